@@ -1,0 +1,429 @@
+"""fp64 CPU oracle for the MuSe (Multipole Semantic Attention) layer.
+
+TEST INFRASTRUCTURE ONLY.  This file is the independent, slow, plain statement
+of what the layer computes, written from the paper.  Only the tests, the smoke
+check and the benchmark's CPU-baseline leg may import it; the CUDA product path
+never does, and the two share no code.  Everything is numpy float64; a library
+matmul / argsort is used as a step, nothing is blocked, fused or reordered.
+
+One (batch, query head) at a time.  Notation follows the paper: queries q,
+keys k, values v, query centroids qbar_i, key clusters j, spatial blocks b of
+size B_s = N / S, per-block summaries (mu, kappa, nu)_{ijb} = (log mass,
+tilted key centroid, tilted value centroid), accumulated (exclusive over
+blocks) summaries (muh, kah, nuh)_{ijb}, k_1 = m retrieved clusters.
+
+Readings taken where the paper is silent (listed again in the design notes):
+ * the softmax scale sigma multiplies every logit: exp(sigma q.k); the paper
+   writes exp(q.k).  qbar is in the units of q, so tilt logits are
+   sigma qbar_i . k and the residual is qres = sigma (q - qbar_i).
+ * clustering: T Lloyd iterations (assign, update) from given start points,
+   then a final assignment against the last centres; qbar := those centres.
+   Empty clusters keep their centre; ties go to the lowest index.
+ * spatial selection k_2 = all causally visible blocks, so the merge has three
+   non-empty components (far approximation, retrieved exact, local exact).
+ * top-m: among clusters with at least one visible key, largest score first,
+   ties to the lower cluster index; fewer than m candidates -> take them all.
+
+Pins (tests/test_oracle_*.py): Lloyd vs scikit-learn / scipy on the same start
+centres; the Algorithm-1 recurrence vs the direct definition of accumulated
+summaries; m = C_k, singleton key clusters or singleton query clusters give
+dense causal softmax attention (textbook formula written separately in the
+test); key-translation invariance; weights sum to one and are causal;
+error bilinear in the residuals; backward vs central finite differences and,
+for m = C_k, vs the closed-form dense-attention gradient.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+__all__ = [
+    "lloyd", "assign_nearest", "assignment_gaps", "strided_init", "feistel_permute",
+    "block_summaries", "accumulate", "accumulated_summaries",
+    "select_clusters", "forward", "backward", "layer_forward", "layer_backward",
+]
+
+_M64 = (1 << 64) - 1
+
+
+# --------------------------------------------------------------------------------------------
+# Clustering (Section "Clustering"; Appendix "Clustering Details")
+# --------------------------------------------------------------------------------------------
+
+def assign_nearest(X, centres):
+    """argmin_c (|c|^2 - 2 x.c): the |x|^2 term cancels between centres
+    (Appendix "Balanced Assignment", distance identity).  Ties -> lowest c."""
+    X = np.asarray(X, np.float64)
+    centres = np.asarray(centres, np.float64)
+    d = (centres * centres).sum(1)[None, :] - 2.0 * (X @ centres.T)
+    return np.argmin(d, axis=1).astype(np.int32)
+
+
+def assignment_gaps(X, centres):
+    """Relative gap (d2 - d1) / max(d2, 1e-30) between the two smallest true squared
+    distances of every point; a point whose gap is below 1e-4 is a near-tie."""
+    X = np.asarray(X, np.float64)
+    centres = np.asarray(centres, np.float64)
+    d = ((X * X).sum(1)[:, None] + (centres * centres).sum(1)[None, :] - 2.0 * (X @ centres.T))
+    d = np.maximum(d, 0.0)
+    if d.shape[1] == 1:
+        return np.ones(d.shape[0])
+    part = np.partition(d, 1, axis=1)
+    d1, d2 = part[:, 0], part[:, 1]
+    return (d2 - d1) / np.maximum(d2, 1e-30)
+
+
+def update_centres(X, a, centres):
+    """Mean of the members of each cluster; an empty cluster keeps its centre."""
+    X = np.asarray(X, np.float64)
+    new = np.array(centres, np.float64, copy=True)
+    for c in range(new.shape[0]):
+        mem = np.nonzero(a == c)[0]
+        if mem.size:
+            new[c] = X[mem].sum(0) / mem.size
+    return new
+
+
+def lloyd(X, T, init_idx=None, init_centres=None):
+    """T x (assign, update) then a final assignment.  Returns (assign, centres)."""
+    X = np.asarray(X, np.float64)
+    centres = (np.array(init_centres, np.float64, copy=True) if init_centres is not None
+               else X[np.asarray(init_idx, np.int64)].copy())
+    for _ in range(T):
+        a = assign_nearest(X, centres)
+        centres = update_centres(X, a, centres)
+    return assign_nearest(X, centres), centres
+
+
+def _splitmix64(x: int) -> int:
+    z = (x + 0x9E3779B97F4A7C15) & _M64
+    z = ((z ^ (z >> 30)) * 0xBF58476D1CE4E5B9) & _M64
+    z = ((z ^ (z >> 27)) * 0x94D049BB133111EB) & _M64
+    return z ^ (z >> 31)
+
+
+def feistel_permute(x: int, N: int, seed: int, stream: int) -> int:
+    """A seeded bijection of [0, N): 4-round balanced Feistel network over the smallest
+    even-width power of two >= N, cycle-walked back into range.  Integer-only, so two
+    independent implementations agree bit for bit."""
+    bits = max(2, (N - 1).bit_length())
+    bits += bits & 1
+    half = bits // 2
+    mask = (1 << half) - 1
+    while True:
+        L, R = x >> half, x & mask
+        for r in range(4):
+            f = _splitmix64((seed ^ (stream << 32) ^ (r << 56) ^ R) & _M64) & mask
+            L, R = R, L ^ f
+        x = (L << half) | R
+        if x < N:
+            return x
+
+
+def strided_init(N: int, C: int, seed: int, stream: int) -> np.ndarray:
+    """Start indices by the paper's rule (Appendix "Centroid Computation", step 1): shuffle
+    with a fixed seed, then take every floor(N/C)-th vector.  The shuffle is the seeded
+    bijection above: index r -> position pi(r * floor(N/C))."""
+    stride = N // C
+    return np.array([feistel_permute(r * stride, N, seed, stream) for r in range(C)], np.int32)
+
+
+# --------------------------------------------------------------------------------------------
+# Summaries (Section "Summary Computation and Causal Accumulation", Eq. 3-5; Algorithm 1)
+# --------------------------------------------------------------------------------------------
+
+def _tilted(qbar, Kmem, Vmem, sigma):
+    """Exact attention from every query centroid to a set of keys: (log mass, key mean, value mean)."""
+    Cq = qbar.shape[0]
+    if Kmem.shape[0] == 0:
+        return (np.full(Cq, -np.inf), np.zeros((Cq, Kmem.shape[1])), np.zeros((Cq, Vmem.shape[1])))
+    l = sigma * (qbar @ Kmem.T)                          # [Cq, n]
+    mx = l.max(1, keepdims=True)
+    w = np.exp(l - mx)
+    s = w.sum(1, keepdims=True)
+    mu = (mx + np.log(s))[:, 0]
+    w = w / s
+    return mu, w @ Kmem, w @ Vmem
+
+
+def block_summaries(K, V, a_k, qbar, sigma, S, Ck):
+    """Per-block summaries of Eq. 3-5: for block b, query cluster i, key cluster j,
+    S_ijb = sum_{k in (b,j)} exp(sigma qbar_i.k); mu = log S; kappa, nu = weighted means.
+    Shapes [S,Cq,Ck], [S,Cq,Ck,D], [S,Cq,Ck,Dv]."""
+    K = np.asarray(K, np.float64); V = np.asarray(V, np.float64); qbar = np.asarray(qbar, np.float64)
+    N, D = K.shape; Dv = V.shape[1]; Cq = qbar.shape[0]; Bs = N // S
+    blk = np.arange(N) // Bs
+    mu = np.full((S, Cq, Ck), -np.inf)
+    kappa = np.zeros((S, Cq, Ck, D)); nu = np.zeros((S, Cq, Ck, Dv))
+    for b in range(S):
+        for j in range(Ck):
+            mem = np.nonzero((blk == b) & (a_k == j))[0]
+            mu[b, :, j], kappa[b, :, j], nu[b, :, j] = _tilted(qbar, K[mem], V[mem], sigma)
+    return mu, kappa, nu
+
+
+def accumulate(mu, kappa, nu):
+    """Exclusive causal accumulation by the recurrence of Algorithm 1:
+    accum_b = accum_{b-1} (+) summary_{b-1}, where (+) adds masses (log-sum-exp of mu)
+    and averages kappa, nu with the masses as weights.  accum_0 is empty."""
+    S = mu.shape[0]
+    muh = np.full_like(mu, -np.inf); kah = np.zeros_like(kappa); nuh = np.zeros_like(nu)
+    for b in range(1, S):
+        a, c = muh[b - 1], mu[b - 1]
+        mx = np.maximum(a, c)
+        safe = np.where(np.isfinite(mx), mx, 0.0)
+        wa, wc = np.exp(a - safe), np.exp(c - safe)      # exp(-inf) = 0 for empty parts
+        tot = wa + wc
+        with np.errstate(divide="ignore", invalid="ignore"):
+            muh[b] = np.where(tot > 0, safe + np.log(tot), -np.inf)
+            fa = np.where(tot > 0, wa / tot, 0.0)[..., None]
+            fc = np.where(tot > 0, wc / tot, 0.0)[..., None]
+        kah[b] = fa * kah[b - 1] + fc * kappa[b - 1]
+        nuh[b] = fa * nuh[b - 1] + fc * nu[b - 1]
+    return muh, kah, nuh
+
+
+def accumulated_summaries(K, V, a_k, qbar, sigma, S, Ck, causal=True):
+    """Accumulated summaries by their direct definition ("accumulated_ijb summarizes all
+    keys/values in blocks 0..b-1 belonging to key cluster j, specialised for query cluster
+    i"): the tilted statistics over M_jb = {u : a_k[u] = j, block(u) < b}.
+    Non-causal: one block whose summary covers every key of the cluster."""
+    K = np.asarray(K, np.float64); V = np.asarray(V, np.float64); qbar = np.asarray(qbar, np.float64)
+    N, D = K.shape; Dv = V.shape[1]; Cq = qbar.shape[0]
+    if not causal:
+        S = 1
+    Bs = N // S
+    blk = np.arange(N) // Bs
+    muh = np.full((S, Cq, Ck), -np.inf)
+    kah = np.zeros((S, Cq, Ck, D)); nuh = np.zeros((S, Cq, Ck, Dv))
+    for b in range(S):
+        for j in range(Ck):
+            vis = (blk < b) if causal else np.ones(N, bool)
+            mem = np.nonzero(vis & (a_k == j))[0]
+            muh[b, :, j], kah[b, :, j], nuh[b, :, j] = _tilted(qbar, K[mem], V[mem], sigma)
+    return muh, kah, nuh
+
+
+# --------------------------------------------------------------------------------------------
+# Per-query attention (Section "Two-Level Retrieval", Eq. 6; "Exact Retrieval and Local
+# Attention"; "Output merging")
+# --------------------------------------------------------------------------------------------
+
+def select_clusters(score, rank_key, m):
+    """Top-m key clusters per row.  `rank_key` [n, Ck] is what is ranked (the Eq. 6 score, or
+    mu alone for per-query-cluster selection); -inf marks clusters with no visible key.
+    Returns int32 [n, m], padded with -1."""
+    n, Ck = rank_key.shape
+    sel = np.full((n, m), -1, np.int32)
+    if m == 0:
+        return sel
+    order = np.argsort(-rank_key, axis=1, kind="stable")      # ties -> lower index
+    for r in range(n):
+        cand = order[r][np.isfinite(rank_key[r, order[r]])][:m]
+        sel[r, :cand.size] = cand
+    return sel
+
+
+def _lse(x, axis):
+    mx = np.max(x, axis=axis, keepdims=True)
+    safe = np.where(np.isfinite(mx), mx, 0.0)
+    with np.errstate(divide="ignore"):
+        out = safe + np.log(np.sum(np.exp(x - safe), axis=axis, keepdims=True))
+    return np.squeeze(out, axis=axis)
+
+
+def _softmax_part(logits, values):
+    """(o, lse) of one component: softmax over the finite logits of each row; rows with no
+    finite logit give lse = -inf and o = 0."""
+    lse = _lse(logits, 1)
+    safe = np.where(np.isfinite(lse), lse, 0.0)
+    p = np.exp(logits - safe[:, None])
+    p[~np.isfinite(lse)] = 0.0
+    return p @ values, lse
+
+
+def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs, m, causal,
+             sel_rows, sel_mode):
+    """All quantities of Algorithm 1's per-query loop for the queries `rows`, which share the
+    query cluster (centroid qbar_i) and the spatial block b."""
+    N = K.shape[0]
+    Ck = muh_ib.shape[0]
+    qp = sigma * Q[rows]                                   # full (scaled) query
+    qres = qp - sigma * qbar_i[None, :]                    # residual
+    score = qres @ kah_ib.T + muh_ib[None, :]              # Eq. 6
+    nonempty = np.isfinite(muh_ib)
+    score = np.where(nonempty[None, :], score, -np.inf)
+    if sel_rows is None:
+        rank = score if sel_mode == 0 else np.broadcast_to(np.where(nonempty, muh_ib, -np.inf), score.shape)
+        sel_rows = select_clusters(score, rank, m)
+    selmask = np.zeros((len(rows), Ck), bool)
+    for r in range(len(rows)):
+        s = sel_rows[r][sel_rows[r] >= 0]
+        selmask[r, s] = True
+    # 1. far field: approximate attention over the clusters that were not retrieved
+    far_logit = np.where(nonempty[None, :] & ~selmask, score, -np.inf)
+    o_far, lse_far = _softmax_part(far_logit, nuh_ib)
+    # 3. exact attention over the retrieved clusters' visible keys (full query)
+    u = np.arange(N)
+    vis = (u // Bs < b) if causal else np.ones(N, bool)
+    ret_mask = vis[None, :] & selmask[:, a_k]
+    logit = qp @ K.T
+    ret_logit = np.where(ret_mask, logit, -np.inf)
+    o_ret, lse_ret = _softmax_part(ret_logit, V)
+    # 4. exact causal attention inside the query's own block
+    if causal:
+        loc_mask = (u[None, :] // Bs == b) & (u[None, :] <= np.asarray(rows)[:, None])
+    else:
+        loc_mask = np.zeros((len(rows), N), bool)
+    loc_logit = np.where(loc_mask, logit, -np.inf)
+    o_loc, lse_loc = _softmax_part(loc_logit, V)
+    # merge by log-sum-exp weights (component 2 is empty because k_2 = all)
+    lses = np.stack([lse_far, lse_ret, lse_loc], 1)
+    L = _lse(lses, 1)
+    wts = np.exp(lses - L[:, None])
+    O = wts[:, 0:1] * o_far + wts[:, 1:2] * o_ret + wts[:, 2:3] * o_loc
+    return dict(O=O, L=L, sel=sel_rows, selmask=selmask, score=score, qp=qp, qres=qres,
+                far_logit=far_logit, exact_logit=np.where(ret_mask | loc_mask, logit, -np.inf),
+                o_far=o_far, lse_far=lse_far, o_ret=o_ret, lse_ret=lse_ret,
+                o_loc=o_loc, lse_loc=lse_loc)
+
+
+def _segments(a_q, N, S, causal, rows):
+    Bs = N // S
+    blk = np.arange(N) // Bs if causal else np.zeros(N, np.int64)
+    keep = np.zeros(N, bool)
+    keep[np.arange(N) if rows is None else np.asarray(rows)] = True
+    for b in range(S if causal else 1):
+        for i in np.unique(a_q[(blk == b) & keep]):
+            yield b, int(i), np.nonzero((blk == b) & (a_q == i) & keep)[0]
+
+
+def forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, sel_mode=0,
+            summ=None, rows=None):
+    """MuSe attention for one head.  Returns a dict with O [N,Dv], LSE [N], sel [N,m] and the
+    three component (o, lse) pairs.  `sel` forces the retrieved clusters (teacher forcing);
+    `rows` restricts the computation to some queries (others are left zero / -inf / -1)."""
+    Q = np.asarray(Q, np.float64); K = np.asarray(K, np.float64); V = np.asarray(V, np.float64)
+    qbar = np.asarray(qbar, np.float64)
+    N, D = Q.shape; Dv = V.shape[1]
+    if not causal:
+        S = 1
+    Bs = N // S
+    if summ is None:
+        summ = accumulated_summaries(K, V, a_k, qbar, sigma, S, Ck, causal)
+    muh, kah, nuh = summ
+    out = dict(O=np.zeros((N, Dv)), LSE=np.full(N, -np.inf), sel=np.full((N, m), -1, np.int32))
+    for name in ("o_far", "o_ret", "o_loc"):
+        out[name] = np.zeros((N, Dv))
+    for name in ("lse_far", "lse_ret", "lse_loc"):
+        out[name] = np.full(N, -np.inf)
+    for b, i, r in _segments(a_q, N, S, causal, rows):
+        seg = _segment(Q, K, V, a_k, qbar[i], muh[b, i], kah[b, i], nuh[b, i], r, b,
+                       sigma=sigma, Bs=Bs, m=m, causal=causal,
+                       sel_rows=None if sel is None else sel[r], sel_mode=sel_mode)
+        out["O"][r], out["LSE"][r], out["sel"][r] = seg["O"], seg["L"], seg["sel"]
+        for name in ("o_far", "lse_far", "o_ret", "lse_ret", "o_loc", "lse_loc"):
+            out[name][r] = seg[name]
+    out["summ"] = summ
+    return out
+
+
+def backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, sel_mode=0,
+             agg_grad=True, rows=None):
+    """Gradients of sum(O * dO) w.r.t. Q, K, V with the assignments, the selections and the
+    query centroids held constant (Appendix "Centroid Gradient Flow"; assignments and
+    selections are discrete).  agg_grad=False also treats the tilted aggregation weights as
+    constants (Appendix "Aggregation Weight Gradient Flow").  Returns (dQ, dK, dV, fwd)."""
+    Q = np.asarray(Q, np.float64); K = np.asarray(K, np.float64); V = np.asarray(V, np.float64)
+    dO = np.asarray(dO, np.float64); qbar = np.asarray(qbar, np.float64)
+    N, D = Q.shape; Dv = V.shape[1]; Cq = qbar.shape[0]
+    if not causal:
+        S = 1
+    Bs = N // S
+    muh, kah, nuh = accumulated_summaries(K, V, a_k, qbar, sigma, S, Ck, causal)
+    dQ = np.zeros((N, D)); dK = np.zeros((N, D)); dV = np.zeros((N, Dv))
+    dmu = np.zeros_like(muh); dka = np.zeros_like(kah); dnu = np.zeros_like(nuh)
+    fwd = dict(O=np.zeros((N, Dv)), LSE=np.full(N, -np.inf), sel=np.full((N, m), -1, np.int32))
+    for b, i, r in _segments(a_q, N, S, causal, rows):
+        seg = _segment(Q, K, V, a_k, qbar[i], muh[b, i], kah[b, i], nuh[b, i], r, b,
+                       sigma=sigma, Bs=Bs, m=m, causal=causal,
+                       sel_rows=None if sel is None else sel[r], sel_mode=sel_mode)
+        fwd["O"][r], fwd["LSE"][r], fwd["sel"][r] = seg["O"], seg["L"], seg["sel"]
+        L = seg["L"][:, None]
+        g_out = dO[r]
+        delta = (g_out * seg["O"]).sum(1, keepdims=True)
+        # the merged output is one softmax over {exact keys} U {far clusters}
+        P = np.exp(seg["exact_logit"] - L)                 # [n, N], zero where masked
+        dV += P.T @ g_out
+        G = P * (g_out @ V.T - delta)
+        dqp = G @ K
+        dK += G.T @ seg["qp"]
+        Pf = np.exp(seg["far_logit"] - L)                  # [n, Ck]
+        dnu[b, i] += Pf.T @ g_out
+        Gf = Pf * (g_out @ nuh[b, i].T - delta)
+        dqp += Gf @ kah[b, i]                              # d score / d q = kah (qbar constant)
+        dka[b, i] += Gf.T @ seg["qres"]
+        dmu[b, i] += Gf.sum(0)
+        dQ[r] = sigma * dqp
+    # through the accumulated summaries to the keys and values they were built from
+    blk = np.arange(N) // Bs
+    for b in range(S):
+        for j in range(Ck):
+            vis = (blk < b) if causal else np.ones(N, bool)
+            mem = np.nonzero(vis & (a_k == j))[0]
+            if mem.size == 0:
+                continue
+            l = sigma * (qbar @ K[mem].T)                  # [Cq, n]
+            w = np.exp(l - muh[b, :, j][:, None])          # normalised tilt weights
+            dK[mem] += w.T @ dka[b, :, j]
+            dV[mem] += w.T @ dnu[b, :, j]
+            if agg_grad:
+                dl = w * (dmu[b, :, j][:, None]
+                          + dka[b, :, j] @ K[mem].T - (dka[b, :, j] * kah[b, :, j]).sum(1)[:, None]
+                          + dnu[b, :, j] @ V[mem].T - (dnu[b, :, j] * nuh[b, :, j]).sum(1)[:, None])
+                dK[mem] += sigma * (dl.T @ qbar)
+    return dQ, dK, dV, fwd
+
+
+# --------------------------------------------------------------------------------------------
+# Whole layer with grouped-query heads: [B,Hq,N,D] queries over [B,Hkv,N,D] keys/values
+# --------------------------------------------------------------------------------------------
+
+def _head_map(Hq, Hkv, head_map):
+    return [h * Hkv // Hq for h in range(Hq)] if head_map is None else list(head_map)
+
+
+def layer_forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, sel_mode=0,
+                  head_map=None):
+    B, Hq, N, D = Q.shape
+    Hkv = K.shape[1]
+    hm = _head_map(Hq, Hkv, head_map)
+    O = np.zeros((B, Hq, N, V.shape[-1])); LSE = np.zeros((B, Hq, N))
+    SEL = np.full((B, Hq, N, m), -1, np.int32)
+    for b in range(B):
+        for h in range(Hq):
+            g = hm[h]
+            f = forward(Q[b, h], K[b, g], V[b, g], a_q[b, h], a_k[b, g], qbar[b, h], sigma=sigma,
+                        S=S, Ck=Ck, m=m, causal=causal, sel=None if sel is None else sel[b, h],
+                        sel_mode=sel_mode)
+            O[b, h], LSE[b, h], SEL[b, h] = f["O"], f["LSE"], f["sel"]
+    return O, LSE, SEL
+
+
+def layer_backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None,
+                   sel_mode=0, agg_grad=True, head_map=None):
+    """dK, dV of a kv head are the sums over the query heads that share it."""
+    B, Hq, N, D = Q.shape
+    Hkv = K.shape[1]
+    hm = _head_map(Hq, Hkv, head_map)
+    dQ = np.zeros(Q.shape); dK = np.zeros(K.shape); dV = np.zeros(V.shape)
+    for b in range(B):
+        for h in range(Hq):
+            g = hm[h]
+            q, k, v, _ = backward(Q[b, h], K[b, g], V[b, g], dO[b, h], a_q[b, h], a_k[b, g],
+                                  qbar[b, h], sigma=sigma, S=S, Ck=Ck, m=m, causal=causal,
+                                  sel=None if sel is None else sel[b, h], sel_mode=sel_mode,
+                                  agg_grad=agg_grad)
+            dQ[b, h] = q
+            dK[b, g] += k
+            dV[b, g] += v
+    return dQ, dK, dV
