@@ -1,0 +1,151 @@
+/*
+ * muse.h — C ABI of the B200 (sm_100a) implementation of the Multipole Semantic Attention
+ * (MuSe) layer: approximate causal softmax attention, forward and backward.
+ *
+ * The four stages follow the paper's Algorithm 1 ("MuSe Causal Attention"):
+ *   muse_cluster    — lines "Cluster Q / Cluster K" (Section "Clustering", Appendix
+ *                     "Clustering Details"), as Lloyd iterations;
+ *   muse_summarize  — "Per-block summaries" and "Causal accumulation along spatial axis"
+ *                     (Section "Summary Computation and Causal Accumulation", Eq. 3-5);
+ *   muse_attn_fwd   — "Two-level retrieval + attention (per query)" and the log-sum-exp merge
+ *                     (Sections "Two-Level Retrieval", Eq. 6, "Exact Retrieval and Local
+ *                     Attention", "Output merging");
+ *   muse_attn_bwd   — gradients with assignments, selections and query centroids held constant
+ *                     (Appendix "Centroid Gradient Flow", "Aggregation Weight Gradient Flow").
+ *
+ * General conventions
+ *   - Every tensor pointer is a DEVICE pointer to a contiguous row-major array unless marked
+ *     HOST.  Q, O, dO, dQ are [B,Hq,N,D]; K, V, dK, dV are [B,Hkv,N,D]; D is innermost.
+ *     Element type is given by muse_params_t.dtype (bf16 or fp32); centroids, LSE and
+ *     summaries are always fp32; indices are int32.
+ *   - The caller owns every buffer.  The library never allocates, frees or synchronises: all
+ *     work is enqueued on `stream` and the call returns at once.  Scratch memory is passed as
+ *     (ws, ws_bytes); sizes come from muse_workspace_bytes.  Workspaces may be reused between
+ *     calls on the same stream.  Pointers must be 16-byte aligned.
+ *   - Return value: MUSE_OK (0) or a negative MUSE_ERR_* code.  Arguments are checked on the
+ *     host before anything is launched; nothing aborts or throws.
+ *   - Spatial blocks: block(t) = t / (N / n_blocks).  Keys are bucketed cluster-major,
+ *     block-minor: bucket (j,b) occupies positions [off_k[j*S+b], off_k[j*S+b+1]) of the
+ *     permutation perm_k (position -> original key index, stable, i.e. ascending inside a
+ *     bucket).
+ */
+#ifndef MUSE_H_
+#define MUSE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#ifndef __DRIVER_TYPES_H__
+typedef struct CUstream_st* cudaStream_t;
+#endif
+
+#if defined(__GNUC__)
+#define MUSE_API __attribute__((visibility("default")))
+#else
+#define MUSE_API
+#endif
+
+enum { MUSE_BF16 = 0, MUSE_F32 = 1 };
+enum { MUSE_SEL_PER_QUERY = 0, MUSE_SEL_PER_QCLUSTER = 1 };
+enum { MUSE_INIT_INDICES = 0, MUSE_INIT_STRIDED = 1, MUSE_INIT_CENTRES = 2 };
+enum {
+  MUSE_OK = 0,
+  MUSE_ERR_INVALID_ARG = -1,   /* null pointer, bad size, misaligned pointer            */
+  MUSE_ERR_UNSUPPORTED = -2,   /* legal request that this build does not implement       */
+  MUSE_ERR_WORKSPACE = -3,     /* ws_bytes smaller than muse_workspace_bytes reports     */
+  MUSE_ERR_CUDA = -4           /* a CUDA runtime call (launch, attribute) failed         */
+};
+
+typedef struct muse_params {
+  int32_t B, Hq, Hkv, N, D;     /* D in {64,128}; Hq % Hkv == 0 unless head_map is given; Hq <= 128 */
+  int32_t Cq, Ck, m;            /* 1 <= Cq <= 4096, 1 <= Ck <= 4096, 0 <= m <= min(Ck,64)          */
+  int32_t causal;               /* 1: blocked causal handling of the paper; 0: one block, no local */
+  int32_t n_blocks;             /* S, spatial blocks (0 -> 8); N % S == 0; forced to 1 if !causal  */
+  int32_t k2;                   /* spatial selection: 0 = all visible blocks (the only value built) */
+  int32_t dtype;                /* MUSE_BF16 | MUSE_F32: type of Q,K,V,O,dO,dQ,dK,dV               */
+  float   softmax_scale;        /* sigma; <= 0 -> 1/sqrt(D)                                        */
+  int32_t kmeans_iters;         /* T Lloyd iterations before the final assignment (>= 0)           */
+  int32_t init_mode;            /* MUSE_INIT_*                                                     */
+  uint64_t seed;                /* used by MUSE_INIT_STRIDED                                       */
+  int32_t sel_mode;             /* MUSE_SEL_*: rank clusters by the Eq. 6 score per query, or by
+                                   the accumulated log-mass per (query cluster, block)            */
+  int32_t dipole;               /* must be 0 (the dipole correction of Appendix B is not built)    */
+  int32_t agg_grad;             /* 1: differentiate the tilted aggregation weights; 0: constants   */
+  const int32_t* head_map;      /* HOST [Hq] -> kv head, or NULL for h * Hkv / Hq                  */
+} muse_params_t;
+
+/* Sizes in bytes of the scratch each stage needs and of the opaque summaries buffer.
+ * out[0] cluster, out[1] summarize, out[2] attn_fwd, out[3] attn_bwd, out[4] summaries.
+ * Appendix "Clustering Cost" / Section "Summary Computation": the summaries buffer holds the
+ * S-1 accumulated (mu, kappa, nu) planes, [B,Hq,S-1,Cq,Ck] x (1 + 2D) fp32, followed by the
+ * bucketed copies of K and V. */
+MUSE_API int muse_workspace_bytes(const muse_params_t* p, size_t out[5]);
+
+/* Byte offsets inside the summaries buffer: off[0] mu [B,Hq,SB,Cq,Ck] f32, off[1] kappa
+ * [B,Hq,SB,Cq,Ck,D] f32, off[2] nu (same), off[3] K bucketed [B,Hkv,N,D] dtype, off[4] V
+ * bucketed; SB = S-1 (causal) or 1.  Plane s of mu/kappa/nu is the accumulated summary seen
+ * by queries of block s+1 (Section "Causal accumulation": exclusive, block 0 sees nothing). */
+MUSE_API int muse_summaries_layout(const muse_params_t* p, size_t off[5]);
+
+/* Lloyd k-means of the queries (per query head, Cq clusters) and keys (per kv head, Ck
+ * clusters): T x (assign to argmin_c |c|^2 - 2 x.c, lowest index on ties; move each centre to
+ * the mean of its members, empty clusters keep theirs), then a final assignment
+ * (Appendix "Clustering Details"; distance identity of "Balanced Assignment").
+ *   Q, K        in   inputs
+ *   init_q/k    in   [B,Hq,Cq] / [B,Hkv,Ck] start indices (MUSE_INIT_INDICES), else NULL
+ *   assign_q/k  out  [B,Hq,N] / [B,Hkv,N] cluster of every query / key
+ *   qbar, kcent out  [B,Hq,Cq,D] / [B,Hkv,Ck,D] fp32 centres used by the final assignment;
+ *                    with MUSE_INIT_CENTRES they are also the input start centres.
+ * Either side may be skipped by passing its Q/K pointer as NULL. */
+MUSE_API int muse_cluster(const muse_params_t* p, const void* Q, const void* K,
+                 const int32_t* init_q, const int32_t* init_k,
+                 int32_t* assign_q, int32_t* assign_k, float* qbar, float* kcent,
+                 void* ws, size_t ws_bytes, cudaStream_t stream);
+
+/* Buckets the keys by (cluster, block) and builds the accumulated tilted summaries
+ * mu_ijb = log sum exp(sigma qbar_i.k), kappa_ijb, nu_ijb = weighted means of k, v over the
+ * keys of cluster j in blocks < b (Eq. 3-5 and "Causal accumulation").
+ *   K, V, assign_k, qbar  in
+ *   off_k     out [B,Hkv,Ck*S+1]   bucket offsets
+ *   perm_k    out [B,Hkv,N]        bucketed position -> key index
+ *   summaries out opaque, muse_workspace_bytes out[4] bytes (layout: muse_summaries_layout) */
+MUSE_API int muse_summarize(const muse_params_t* p, const void* K, const void* V,
+                   const int32_t* assign_k, const float* qbar,
+                   int32_t* off_k, int32_t* perm_k, void* summaries,
+                   void* ws, size_t ws_bytes, cudaStream_t stream);
+
+/* Forward: per query, score every key cluster (Eq. 6), retrieve the top-m for exact
+ * attention, approximate the rest with the summaries, add exact causal attention inside the
+ * query's block, merge by log-sum-exp.
+ *   sel_in   in   [B,Hq,N,m] clusters to retrieve (-1 = none) or NULL to select here
+ *   O        out  [B,Hq,N,D] dtype
+ *   LSE      out  [B,Hq,N] fp32 log of the merged normaliser
+ *   sel_out  out  [B,Hq,N,m] retrieved clusters, best first, padded with -1 (may be NULL) */
+MUSE_API int muse_attn_fwd(const muse_params_t* p, const void* Q, const void* K, const void* V,
+                  const int32_t* assign_q, const float* qbar,
+                  const int32_t* off_k, const int32_t* perm_k, const void* summaries,
+                  const int32_t* sel_in, void* O, float* LSE, int32_t* sel_out,
+                  void* ws, size_t ws_bytes, cudaStream_t stream);
+
+/* Backward of sum(O * dO) w.r.t. Q, K, V with assign_*, sel and qbar constant; dK, dV of a
+ * kv head are summed over the query heads that share it.
+ *   O, LSE, sel  in   as returned by muse_attn_fwd (sel must be the selection used there)
+ *   dQ, dK, dV   out  dtype */
+MUSE_API int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K, const void* V,
+                  const void* O, const float* LSE, const void* dO,
+                  const int32_t* assign_q, const float* qbar,
+                  const int32_t* off_k, const int32_t* perm_k, const void* summaries,
+                  const int32_t* sel, void* dQ, void* dK, void* dV,
+                  void* ws, size_t ws_bytes, cudaStream_t stream);
+
+/* Human-readable text for a return code (static storage). */
+MUSE_API const char* muse_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MUSE_H_ */

@@ -252,9 +252,16 @@ def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs
     score = qres @ kah_ib.T + muh_ib[None, :]              # Eq. 6
     nonempty = np.isfinite(muh_ib)
     score = np.where(nonempty[None, :], score, -np.inf)
+    rank = score if sel_mode == 0 else np.broadcast_to(np.where(nonempty, muh_ib, -np.inf), score.shape)
     if sel_rows is None:
-        rank = score if sel_mode == 0 else np.broadcast_to(np.where(nonempty, muh_ib, -np.inf), score.shape)
         sel_rows = select_clusters(score, rank, m)
+    # diagnostic only: margin between the m-th and (m+1)-th ranked cluster (inf if no choice)
+    srt = -np.sort(-rank, axis=1)
+    if 0 < m < Ck:
+        with np.errstate(invalid="ignore"):
+            gap = np.where(np.isfinite(srt[:, m]), srt[:, m - 1] - srt[:, m], np.inf)
+    else:
+        gap = np.full(len(rows), np.inf)
     selmask = np.zeros((len(rows), Ck), bool)
     for r in range(len(rows)):
         s = sel_rows[r][sel_rows[r] >= 0]
@@ -281,7 +288,7 @@ def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs
     L = _lse(lses, 1)
     wts = np.exp(lses - L[:, None])
     O = wts[:, 0:1] * o_far + wts[:, 1:2] * o_ret + wts[:, 2:3] * o_loc
-    return dict(O=O, L=L, sel=sel_rows, selmask=selmask, score=score, qp=qp, qres=qres,
+    return dict(O=O, L=L, sel=sel_rows, sel_gap=gap, selmask=selmask, score=score, qp=qp, qres=qres,
                 far_logit=far_logit, exact_logit=np.where(ret_mask | loc_mask, logit, -np.inf),
                 o_far=o_far, lse_far=lse_far, o_ret=o_ret, lse_ret=lse_ret,
                 o_loc=o_loc, lse_loc=lse_loc)
@@ -311,7 +318,8 @@ def forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, 
     if summ is None:
         summ = accumulated_summaries(K, V, a_k, qbar, sigma, S, Ck, causal)
     muh, kah, nuh = summ
-    out = dict(O=np.zeros((N, Dv)), LSE=np.full(N, -np.inf), sel=np.full((N, m), -1, np.int32))
+    out = dict(O=np.zeros((N, Dv)), LSE=np.full(N, -np.inf), sel=np.full((N, m), -1, np.int32),
+               sel_gap=np.full(N, np.inf))
     for name in ("o_far", "o_ret", "o_loc"):
         out[name] = np.zeros((N, Dv))
     for name in ("lse_far", "lse_ret", "lse_loc"):
@@ -321,6 +329,7 @@ def forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, 
                        sigma=sigma, Bs=Bs, m=m, causal=causal,
                        sel_rows=None if sel is None else sel[r], sel_mode=sel_mode)
         out["O"][r], out["LSE"][r], out["sel"][r] = seg["O"], seg["L"], seg["sel"]
+        out["sel_gap"][r] = seg["sel_gap"]
         for name in ("o_far", "lse_far", "o_ret", "lse_ret", "o_loc", "lse_loc"):
             out[name][r] = seg[name]
     out["summ"] = summ

@@ -1,0 +1,199 @@
+"""Thin ctypes binding of libmuse.so: argument marshalling only.
+
+Function names and argument order mirror include/muse.h.  Tensors are torch CUDA tensors
+(torch is used for device memory and streams only); every step of the computation runs in
+the library's CUDA kernels.  There is no CPU fallback: a missing library raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmuse.so")
+
+MUSE_BF16, MUSE_F32 = 0, 1
+MUSE_SEL_PER_QUERY, MUSE_SEL_PER_QCLUSTER = 0, 1
+MUSE_INIT_INDICES, MUSE_INIT_STRIDED, MUSE_INIT_CENTRES = 0, 1, 2
+
+EXPORTS = ("muse_workspace_bytes", "muse_summaries_layout", "muse_cluster", "muse_summarize",
+           "muse_attn_fwd", "muse_attn_bwd", "muse_strerror")
+
+
+class MuseParams(ctypes.Structure):
+    """Mirror of muse_params_t."""
+    _fields_ = [
+        ("B", ctypes.c_int32), ("Hq", ctypes.c_int32), ("Hkv", ctypes.c_int32), ("N", ctypes.c_int32),
+        ("D", ctypes.c_int32), ("Cq", ctypes.c_int32), ("Ck", ctypes.c_int32), ("m", ctypes.c_int32),
+        ("causal", ctypes.c_int32), ("n_blocks", ctypes.c_int32), ("k2", ctypes.c_int32),
+        ("dtype", ctypes.c_int32), ("softmax_scale", ctypes.c_float), ("kmeans_iters", ctypes.c_int32),
+        ("init_mode", ctypes.c_int32), ("seed", ctypes.c_uint64), ("sel_mode", ctypes.c_int32),
+        ("dipole", ctypes.c_int32), ("agg_grad", ctypes.c_int32), ("head_map", ctypes.POINTER(ctypes.c_int32)),
+    ]
+
+    @property
+    def S(self) -> int:
+        return (self.n_blocks or 8) if self.causal else 1
+
+    @property
+    def SB(self) -> int:
+        return self.S - 1 if self.causal else 1
+
+    @property
+    def sigma(self) -> float:
+        return self.softmax_scale if self.softmax_scale > 0 else 1.0 / math.sqrt(self.D)
+
+
+def make_params(*, B, Hq, Hkv, N, D, Cq, Ck, m, causal=True, n_blocks=8, dtype="bf16", softmax_scale=0.0,
+                kmeans_iters=3, init_mode=MUSE_INIT_INDICES, seed=0, sel_mode=MUSE_SEL_PER_QUERY,
+                agg_grad=True, head_map=None, k2=0, dipole=0) -> MuseParams:
+    p = MuseParams(B=B, Hq=Hq, Hkv=Hkv, N=N, D=D, Cq=Cq, Ck=Ck, m=m, causal=int(causal), n_blocks=n_blocks,
+                   k2=k2, dtype=MUSE_F32 if dtype in ("f32", torch.float32) else MUSE_BF16,
+                   softmax_scale=softmax_scale, kmeans_iters=kmeans_iters, init_mode=init_mode, seed=seed,
+                   sel_mode=sel_mode, dipole=dipole, agg_grad=int(agg_grad))
+    if head_map is not None:
+        arr = (ctypes.c_int32 * Hq)(*[int(x) for x in head_map])
+        p._head_map_keepalive = arr
+        p.head_map = ctypes.cast(arr, ctypes.POINTER(ctypes.c_int32))
+    return p
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Loads libmuse.so (once).  Raises if it has not been built: there is no fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2509_10406_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i32p, f32p, sz = ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t
+        pp = ctypes.POINTER(MuseParams)
+        L.muse_strerror.restype = ctypes.c_char_p
+        L.muse_strerror.argtypes = [ctypes.c_int]
+        L.muse_workspace_bytes.argtypes = [pp, ctypes.POINTER(sz)]
+        L.muse_summaries_layout.argtypes = [pp, ctypes.POINTER(sz)]
+        L.muse_cluster.argtypes = [pp, vp, vp, i32p, i32p, i32p, i32p, f32p, f32p, vp, sz, vp]
+        L.muse_summarize.argtypes = [pp, vp, vp, i32p, f32p, i32p, i32p, vp, vp, sz, vp]
+        L.muse_attn_fwd.argtypes = [pp, vp, vp, vp, i32p, f32p, i32p, i32p, vp, i32p, vp, f32p, i32p, vp, sz, vp]
+        L.muse_attn_bwd.argtypes = [pp, vp, vp, vp, vp, f32p, vp, i32p, f32p, i32p, i32p, vp, i32p, vp, vp, vp,
+                                    vp, sz, vp]
+        for name in EXPORTS[:-1]:
+            getattr(L, name).restype = ctypes.c_int
+        _lib = L
+    return _lib
+
+
+class MuseError(RuntimeError):
+    pass
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        raise MuseError(f"{what}: {lib().muse_strerror(rc).decode()} ({rc})")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "tensors must be contiguous CUDA tensors"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def muse_workspace_bytes(p: MuseParams):
+    """(cluster, summarize, attn_fwd, attn_bwd, summaries) sizes in bytes."""
+    out = (ctypes.c_size_t * 5)()
+    _check(lib().muse_workspace_bytes(ctypes.byref(p), out), "muse_workspace_bytes")
+    return tuple(int(x) for x in out)
+
+
+def muse_summaries_layout(p: MuseParams):
+    out = (ctypes.c_size_t * 5)()
+    _check(lib().muse_summaries_layout(ctypes.byref(p), out), "muse_summaries_layout")
+    return tuple(int(x) for x in out)
+
+
+def muse_cluster(p, Q, K, init_q, init_k, assign_q, assign_k, qbar, kcent, ws):
+    _check(lib().muse_cluster(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(init_q), _ptr(init_k), _ptr(assign_q),
+                              _ptr(assign_k), _ptr(qbar), _ptr(kcent), _ptr(ws), ws.numel() * ws.element_size(),
+                              _stream()), "muse_cluster")
+
+
+def muse_summarize(p, K, V, assign_k, qbar, off_k, perm_k, summaries, ws):
+    _check(lib().muse_summarize(ctypes.byref(p), _ptr(K), _ptr(V), _ptr(assign_k), _ptr(qbar), _ptr(off_k),
+                                _ptr(perm_k), _ptr(summaries), _ptr(ws), ws.numel() * ws.element_size(),
+                                _stream()), "muse_summarize")
+
+
+def muse_attn_fwd(p, Q, K, V, assign_q, qbar, off_k, perm_k, summaries, sel_in, O, LSE, sel_out, ws):
+    _check(lib().muse_attn_fwd(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(assign_q), _ptr(qbar), _ptr(off_k),
+                               _ptr(perm_k), _ptr(summaries), _ptr(sel_in), _ptr(O), _ptr(LSE), _ptr(sel_out),
+                               _ptr(ws), ws.numel() * ws.element_size(), _stream()), "muse_attn_fwd")
+
+
+def muse_attn_bwd(p, Q, K, V, O, LSE, dO, assign_q, qbar, off_k, perm_k, summaries, sel, dQ, dK, dV, ws):
+    _check(lib().muse_attn_bwd(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(LSE), _ptr(dO),
+                               _ptr(assign_q), _ptr(qbar), _ptr(off_k), _ptr(perm_k), _ptr(summaries), _ptr(sel),
+                               _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
+           "muse_attn_bwd")
+
+
+# ---------------------------------------------------------------------------------------------
+# Buffer plumbing (allocation only)
+# ---------------------------------------------------------------------------------------------
+
+class MuseBuffers:
+    """Owns the device buffers one layer call needs (outputs, intermediates, workspaces)."""
+
+    def __init__(self, p: MuseParams, device="cuda", backward=True):
+        self.p = p
+        dt = torch.float32 if p.dtype == MUSE_F32 else torch.bfloat16
+        i32, f32 = torch.int32, torch.float32
+        B, Hq, Hkv, N, D, m = p.B, p.Hq, p.Hkv, p.N, p.D, p.m
+        sizes = muse_workspace_bytes(p)
+        e = lambda *s, dtype: torch.empty(*s, dtype=dtype, device=device)
+        self.assign_q = e(B, Hq, N, dtype=i32); self.assign_k = e(B, Hkv, N, dtype=i32)
+        self.qbar = e(B, Hq, p.Cq, D, dtype=f32); self.kcent = e(B, Hkv, p.Ck, D, dtype=f32)
+        self.off_k = e(B, Hkv, p.Ck * p.S + 1, dtype=i32); self.perm_k = e(B, Hkv, N, dtype=i32)
+        self.summaries = e(sizes[4], dtype=torch.uint8)
+        self.O = e(B, Hq, N, D, dtype=dt); self.LSE = e(B, Hq, N, dtype=f32)
+        self.sel = e(B, Hq, N, max(m, 1), dtype=i32)
+        need = max(sizes[:3] + ((sizes[3],) if backward else ()))
+        self.ws = e(need, dtype=torch.uint8)
+        if backward:
+            self.dQ = e(B, Hq, N, D, dtype=dt); self.dK = e(B, Hkv, N, D, dtype=dt); self.dV = e(B, Hkv, N, D, dtype=dt)
+
+    def summary_planes(self):
+        """Views (mu, kappa, nu) of the accumulated summaries: [B,Hq,SB,Cq,Ck(,D)] fp32."""
+        p = self.p
+        off = muse_summaries_layout(p)
+        ent = p.B * p.Hq * p.SB * p.Cq * p.Ck
+        f = lambda o, n: self.summaries[o:o + 4 * n].view(torch.float32)
+        mu = f(off[0], ent).view(p.B, p.Hq, p.SB, p.Cq, p.Ck)
+        ka = f(off[1], ent * p.D).view(p.B, p.Hq, p.SB, p.Cq, p.Ck, p.D)
+        nu = f(off[2], ent * p.D).view(p.B, p.Hq, p.SB, p.Cq, p.Ck, p.D)
+        return mu, ka, nu
+
+
+def muse_layer_forward(p, buf: MuseBuffers, Q, K, V, init_q=None, init_k=None, sel_in=None):
+    """cluster -> summarize -> attention forward on the current stream."""
+    muse_cluster(p, Q, K, init_q, init_k, buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, buf.ws)
+    muse_summarize(p, K, V, buf.assign_k, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
+    muse_attn_fwd(p, Q, K, V, buf.assign_q, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, sel_in, buf.O, buf.LSE,
+                  buf.sel, buf.ws)
+    return buf.O
+
+
+def muse_layer_backward(p, buf: MuseBuffers, Q, K, V, dO, sel=None):
+    muse_attn_bwd(p, Q, K, V, buf.O, buf.LSE, dO, buf.assign_q, buf.qbar, buf.off_k, buf.perm_k, buf.summaries,
+                  buf.sel if sel is None else sel, buf.dQ, buf.dK, buf.dV, buf.ws)
+    return buf.dQ, buf.dK, buf.dV

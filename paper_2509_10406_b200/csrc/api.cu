@@ -1,0 +1,155 @@
+// C-ABI entry points: argument validation on the host, then the stage launchers.
+#include "common.cuh"
+
+using namespace muse;
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Validates the parameter block and resolves defaults.  Returns MUSE_OK or an error code.
+int resolve(const muse_params_t* p, Dims* d) {
+  if (p == nullptr) return MUSE_ERR_INVALID_ARG;
+  if (p->B < 1 || p->Hq < 1 || p->Hkv < 1 || p->N < 1) return MUSE_ERR_INVALID_ARG;
+  if (p->Cq < 1 || p->Ck < 1 || p->m < 0 || p->m > p->Ck) return MUSE_ERR_INVALID_ARG;
+  if (p->Cq > p->N || p->Ck > p->N) return MUSE_ERR_INVALID_ARG;
+  if (p->dtype != MUSE_BF16 && p->dtype != MUSE_F32) return MUSE_ERR_INVALID_ARG;
+  if (p->kmeans_iters < 0 || p->init_mode < 0 || p->init_mode > 2) return MUSE_ERR_INVALID_ARG;
+  if (p->sel_mode != MUSE_SEL_PER_QUERY && p->sel_mode != MUSE_SEL_PER_QCLUSTER) return MUSE_ERR_INVALID_ARG;
+  if (p->n_blocks < 0 || p->k2 < 0) return MUSE_ERR_INVALID_ARG;
+  if (p->D != 64 && p->D != 128) return MUSE_ERR_UNSUPPORTED;
+  if (p->Hq > kMaxHeads || p->m > kMaxM || p->Cq > kMaxC || p->Ck > kMaxC) return MUSE_ERR_UNSUPPORTED;
+  if (p->k2 != 0 || p->dipole != 0) return MUSE_ERR_UNSUPPORTED;
+  int S = p->causal ? (p->n_blocks == 0 ? 8 : p->n_blocks) : 1;
+  if (p->N % S != 0) return MUSE_ERR_INVALID_ARG;
+  if ((long long)S * p->Cq > 32768 || (long long)S * p->Ck > 32768) return MUSE_ERR_UNSUPPORTED;
+  if ((long long)p->N * (p->m > 0 ? p->m : 1) > 0x7fffffffLL) return MUSE_ERR_UNSUPPORTED;
+  d->B = p->B; d->Hq = p->Hq; d->Hkv = p->Hkv; d->N = p->N; d->D = p->D;
+  d->Cq = p->Cq; d->Ck = p->Ck; d->m = p->m;
+  d->S = S; d->SB = p->causal ? S - 1 : 1; d->Bs = p->N / S;
+  d->causal = p->causal ? 1 : 0; d->sel_mode = p->sel_mode; d->agg_grad = p->agg_grad ? 1 : 0;
+  d->sigma = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->D);
+  for (int h = 0; h < kMaxHeads; ++h) d->hm.g[h] = 0;
+  for (int h = 0; h < p->Hq; ++h) {
+    int g;
+    if (p->head_map) g = p->head_map[h];
+    else { if (p->Hq % p->Hkv != 0) return MUSE_ERR_INVALID_ARG; g = (int)((long long)h * p->Hkv / p->Hq); }
+    if (g < 0 || g >= p->Hkv) return MUSE_ERR_INVALID_ARG;
+    d->hm.g[h] = (int16_t)g;
+  }
+  return MUSE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* muse_strerror(int code) {
+  switch (code) {
+    case MUSE_OK: return "ok";
+    case MUSE_ERR_INVALID_ARG: return "invalid argument";
+    case MUSE_ERR_UNSUPPORTED: return "unsupported configuration";
+    case MUSE_ERR_WORKSPACE: return "workspace too small";
+    case MUSE_ERR_CUDA: return "CUDA runtime error";
+    default: return "unknown error";
+  }
+}
+
+int muse_workspace_bytes(const muse_params_t* p, size_t out[5]) {
+  Dims d;
+  int rc = resolve(p, &d);
+  if (rc != MUSE_OK) return rc;
+  if (out == nullptr) return MUSE_ERR_INVALID_ARG;
+  size_t cq = lloyd_ws_bytes(d, d.B * d.Hq, d.Cq, 0), ck = lloyd_ws_bytes(d, d.B * d.Hkv, d.Ck, 1);
+  out[0] = cq > ck ? cq : ck;
+  out[1] = summarize_ws_bytes(d);
+  out[2] = attn_fwd_ws_bytes(d, p->dtype);
+  out[3] = attn_bwd_ws_bytes(d, p->dtype);
+  out[4] = summ_layout(d, p->dtype).total;
+  for (int k = 0; k < 4; ++k) if (out[k] < 256) out[k] = 256;
+  return MUSE_OK;
+}
+
+int muse_summaries_layout(const muse_params_t* p, size_t off[5]) {
+  Dims d;
+  int rc = resolve(p, &d);
+  if (rc != MUSE_OK) return rc;
+  if (off == nullptr) return MUSE_ERR_INVALID_ARG;
+  SummLayout L = summ_layout(d, p->dtype);
+  off[0] = L.mu; off[1] = L.kappa; off[2] = L.nu; off[3] = L.Kp; off[4] = L.Vp;
+  return MUSE_OK;
+}
+
+int muse_cluster(const muse_params_t* p, const void* Q, const void* K, const int32_t* init_q,
+                 const int32_t* init_k, int32_t* assign_q, int32_t* assign_k, float* qbar, float* kcent,
+                 void* ws, size_t ws_bytes, cudaStream_t stream) {
+  Dims d;
+  int rc = resolve(p, &d);
+  if (rc != MUSE_OK) return rc;
+  if (ws == nullptr || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;
+  if (Q == nullptr && K == nullptr) return MUSE_ERR_INVALID_ARG;
+  size_t need[5];
+  muse_workspace_bytes(p, need);
+  if (ws_bytes < need[0]) return MUSE_ERR_WORKSPACE;
+  if (Q != nullptr) {
+    if (assign_q == nullptr || qbar == nullptr || !aligned16(Q) || !aligned16(qbar)) return MUSE_ERR_INVALID_ARG;
+    if (p->init_mode == MUSE_INIT_INDICES && init_q == nullptr) return MUSE_ERR_INVALID_ARG;
+    rc = lloyd(d, p->dtype, Q, d.B * d.Hq, d.Cq, 0, init_q, p->init_mode, p->seed, p->kmeans_iters, assign_q, qbar, ws, stream);
+    if (rc != MUSE_OK) return rc;
+  }
+  if (K != nullptr) {
+    if (assign_k == nullptr || kcent == nullptr || !aligned16(K) || !aligned16(kcent)) return MUSE_ERR_INVALID_ARG;
+    if (p->init_mode == MUSE_INIT_INDICES && init_k == nullptr) return MUSE_ERR_INVALID_ARG;
+    rc = lloyd(d, p->dtype, K, d.B * d.Hkv, d.Ck, 1, init_k, p->init_mode, p->seed, p->kmeans_iters, assign_k, kcent, ws, stream);
+    if (rc != MUSE_OK) return rc;
+  }
+  return MUSE_OK;
+}
+
+int muse_summarize(const muse_params_t* p, const void* K, const void* V, const int32_t* assign_k,
+                   const float* qbar, int32_t* off_k, int32_t* perm_k, void* summaries, void* ws,
+                   size_t ws_bytes, cudaStream_t stream) {
+  Dims d;
+  int rc = resolve(p, &d);
+  if (rc != MUSE_OK) return rc;
+  if (!K || !V || !assign_k || !qbar || !off_k || !perm_k || !summaries || !ws) return MUSE_ERR_INVALID_ARG;
+  if (!aligned16(K) || !aligned16(V) || !aligned16(qbar) || !aligned16(summaries) || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;
+  size_t need[5];
+  muse_workspace_bytes(p, need);
+  if (ws_bytes < need[1]) return MUSE_ERR_WORKSPACE;
+  return summarize(d, p->dtype, K, V, assign_k, qbar, off_k, perm_k, summaries, ws, stream);
+}
+
+int muse_attn_fwd(const muse_params_t* p, const void* Q, const void* K, const void* V,
+                  const int32_t* assign_q, const float* qbar, const int32_t* off_k, const int32_t* perm_k,
+                  const void* summaries, const int32_t* sel_in, void* O, float* LSE, int32_t* sel_out,
+                  void* ws, size_t ws_bytes, cudaStream_t stream) {
+  Dims d;
+  int rc = resolve(p, &d);
+  if (rc != MUSE_OK) return rc;
+  if (!Q || !K || !V || !assign_q || !qbar || !off_k || !perm_k || !summaries || !O || !LSE || !ws) return MUSE_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(qbar) || !aligned16(summaries) || !aligned16(O) || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;
+  size_t need[5];
+  muse_workspace_bytes(p, need);
+  if (ws_bytes < need[2]) return MUSE_ERR_WORKSPACE;
+  return attn_fwd(d, p->dtype, Q, K, V, assign_q, qbar, off_k, perm_k, summaries, sel_in, O, LSE, sel_out, ws, stream);
+}
+
+int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K, const void* V, const void* O,
+                  const float* LSE, const void* dO, const int32_t* assign_q, const float* qbar,
+                  const int32_t* off_k, const int32_t* perm_k, const void* summaries, const int32_t* sel,
+                  void* dQ, void* dK, void* dV, void* ws, size_t ws_bytes, cudaStream_t stream) {
+  Dims d;
+  int rc = resolve(p, &d);
+  if (rc != MUSE_OK) return rc;
+  if (!Q || !K || !V || !O || !LSE || !dO || !assign_q || !qbar || !off_k || !perm_k || !summaries || !dQ || !dK || !dV || !ws) return MUSE_ERR_INVALID_ARG;
+  if (d.m > 0 && d.SB > 0 && sel == nullptr) return MUSE_ERR_INVALID_ARG;
+  if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(qbar) ||
+      !aligned16(summaries) || !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;
+  size_t need[5];
+  muse_workspace_bytes(p, need);
+  if (ws_bytes < need[3]) return MUSE_ERR_WORKSPACE;
+  return attn_bwd(d, p->dtype, Q, K, V, O, LSE, dO, assign_q, qbar, off_k, perm_k, summaries, sel, dQ, dK, dV, ws, stream);
+}
+
+}  // extern "C"

@@ -1,0 +1,361 @@
+// Clustering stage: Lloyd k-means (Appendix "Clustering Details") and the stable
+// (cluster, block) bucketing used by every later stage (Section "Exact retrieval": keys and
+// values are bucketed by (cluster, block)).
+#include "common.cuh"
+
+namespace muse {
+
+// ---------------------------------------------------------------------------------------------
+// Stable counting sort of tokens by an integer key.
+//   kind 0 (queries): key = block * C + cluster   -> segments (block, cluster) contiguous
+//   kind 1 (keys)   : key = cluster * S + block   -> a cluster's blocks are one contiguous run
+// Three kernels: per-chunk histogram, one scan per problem, stable scatter.
+// ---------------------------------------------------------------------------------------------
+constexpr int kSortChunk = 4096;
+constexpr int kSortThreads = 256;
+
+__device__ __forceinline__ int sort_key(int t, int a, int C, int S, int Bs, int kind) {
+  int b = t / Bs;
+  return kind == 0 ? b * C + a : a * S + b;
+}
+
+__global__ void __launch_bounds__(kSortThreads)
+k_sort_hist(const int32_t* __restrict__ assign, int N, int C, int S, int Bs, int kind, int nkeys,
+            int nchunks, int32_t* __restrict__ cnt) {
+  extern __shared__ int32_t sh[];
+  const int chunk = blockIdx.x, prob = blockIdx.y;
+  for (int k = threadIdx.x; k < nkeys; k += kSortThreads) sh[k] = 0;
+  __syncthreads();
+  const int32_t* a = assign + (size_t)prob * N;
+  const int t0 = chunk * kSortChunk, t1 = min(N, t0 + kSortChunk);
+  for (int t = t0 + threadIdx.x; t < t1; t += kSortThreads)
+    atomicAdd(&sh[sort_key(t, a[t], C, S, Bs, kind)], 1);
+  __syncthreads();
+  int32_t* c = cnt + (size_t)prob * nkeys * nchunks;
+  for (int k = threadIdx.x; k < nkeys; k += kSortThreads) c[(size_t)k * nchunks + chunk] = sh[k];
+}
+
+// Exclusive scan of cnt[key][chunk] in (key, chunk) order; off[key] = start of the key's run.
+__global__ void __launch_bounds__(1024)
+k_sort_scan(int32_t* __restrict__ cnt, int nkeys, int nchunks, int32_t* __restrict__ off) {
+  __shared__ int32_t part[1024];
+  const int prob = blockIdx.x, tid = threadIdx.x;
+  const int L = nkeys * nchunks;
+  int32_t* c = cnt + (size_t)prob * L;
+  int32_t* o = off + (size_t)prob * (nkeys + 1);
+  const int per = cdiv(L, 1024);
+  const int e0 = min(L, tid * per), e1 = min(L, e0 + per);
+  int s = 0;
+  for (int e = e0; e < e1; ++e) s += c[e];
+  part[tid] = s;
+  __syncthreads();
+  for (int ofs = 1; ofs < 1024; ofs <<= 1) {       // Hillis-Steele inclusive scan
+    int v = tid >= ofs ? part[tid - ofs] : 0;
+    __syncthreads();
+    part[tid] += v;
+    __syncthreads();
+  }
+  int run = part[tid] - s;
+  for (int e = e0; e < e1; ++e) {
+    int v = c[e];
+    c[e] = run;
+    if (e % nchunks == 0) o[e / nchunks] = run;
+    run += v;
+  }
+  if (tid == 1023) o[nkeys] = run;     // the last thread ends on the grand total
+}
+
+int launch_scan(int32_t* cnt, int problems, int nkeys, int nchunks, int32_t* off, cudaStream_t st) {
+  k_sort_scan<<<problems, 1024, 0, st>>>(cnt, nkeys, nchunks, off);
+  MUSE_LAUNCH_OK();
+  return MUSE_OK;
+}
+
+__global__ void __launch_bounds__(kSortThreads)
+k_sort_scatter(const int32_t* __restrict__ assign, int N, int C, int S, int Bs, int kind, int nkeys,
+               int nchunks, const int32_t* __restrict__ cnt, int32_t* __restrict__ perm) {
+  extern __shared__ int32_t cur[];
+  const int chunk = blockIdx.x, prob = blockIdx.y;
+  const int32_t* c = cnt + (size_t)prob * nkeys * nchunks;
+  for (int k = threadIdx.x; k < nkeys; k += kSortThreads) cur[k] = c[(size_t)k * nchunks + chunk];
+  __syncthreads();
+  const int32_t* a = assign + (size_t)prob * N;
+  int32_t* pm = perm + (size_t)prob * N;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int t0 = chunk * kSortChunk, t1 = min(N, t0 + kSortChunk);
+  for (int base = t0; base < t1; base += kSortThreads) {
+    const int t = base + threadIdx.x;
+    const bool live = t < t1;
+    const int key = live ? sort_key(t, a[t], C, S, Bs, kind) : -1 - lane;
+    // warps take turns in token order so equal keys keep ascending positions (stable)
+    for (int w = 0; w < kSortThreads / 32; ++w) {
+      if (warp == w) {
+        unsigned peers = __match_any_sync(0xffffffffu, key);
+        int rank = __popc(peers & ((1u << lane) - 1u));
+        int start = live ? cur[key] : 0;
+        __syncwarp();
+        if (live) {
+          pm[start + rank] = t;
+          if (rank == __popc(peers) - 1) cur[key] = start + rank + 1;
+        }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+size_t sort_ws_elems(int N, int nkeys) { return (size_t)nkeys * cdiv(N, kSortChunk); }
+
+int bucket_sort(int, const int32_t* assign, int problems, int N, int C, int S, int Bs, int kind,
+                int32_t* off, int32_t* perm, int32_t* scratch, cudaStream_t st) {
+  const int nkeys = C * S, nchunks = cdiv(N, kSortChunk);
+  const size_t smem = (size_t)nkeys * sizeof(int32_t);
+  if (smem > 48 * 1024) {
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_sort_hist, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_sort_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  }
+  k_sort_hist<<<dim3(nchunks, problems), kSortThreads, smem, st>>>(assign, N, C, S, Bs, kind, nkeys, nchunks, scratch);
+  MUSE_LAUNCH_OK();
+  if (launch_scan(scratch, problems, nkeys, nchunks, off, st) != MUSE_OK) return MUSE_ERR_CUDA;
+  k_sort_scatter<<<dim3(nchunks, problems), kSortThreads, smem, st>>>(assign, N, C, S, Bs, kind, nkeys, nchunks, scratch, perm);
+  MUSE_LAUNCH_OK();
+  return MUSE_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Lloyd iterations
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t splitmix64(uint64_t x) {
+  uint64_t z = x + 0x9E3779B97F4A7C15ull;
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
+// Seeded bijection of [0, N): 4-round Feistel network on the smallest even-width power of two
+// that covers N, cycle-walked into range (the "shuffle with a fixed random seed" of Appendix
+// "Centroid Computation", step 1).
+__device__ int feistel_permute(int x0, int N, uint64_t seed, uint64_t stream) {
+  int bits = 32 - __clz(max(N - 1, 1));
+  if (bits < 2) bits = 2;
+  bits += bits & 1;
+  const int half = bits / 2;
+  const uint64_t mask = (1ull << half) - 1ull;
+  uint64_t x = (uint64_t)x0;
+  for (int guard = 0; guard < 1 << 20; ++guard) {
+    uint64_t L = x >> half, R = x & mask;
+#pragma unroll
+    for (uint64_t r = 0; r < 4; ++r) {
+      uint64_t f = splitmix64(seed ^ (stream << 32) ^ (r << 56) ^ R) & mask;
+      uint64_t nl = R; R = L ^ f; L = nl;
+    }
+    x = (L << half) | R;
+    if (x < (uint64_t)N) break;
+  }
+  return (int)x;
+}
+
+template <class T>
+__global__ void k_init_centres(const T* __restrict__ X, int N, int D, int C, const int32_t* __restrict__ init_idx,
+                               int init_mode, uint64_t seed, int kind, float* __restrict__ centres) {
+  const int c = blockIdx.x, prob = blockIdx.y;
+  int idx;
+  if (init_mode == MUSE_INIT_INDICES) idx = init_idx[(size_t)prob * C + c];
+  else idx = feistel_permute(c * (N / C), N, seed, (uint64_t)prob * 2 + kind);
+  idx = min(max(idx, 0), N - 1);
+  const T* x = X + ((size_t)prob * N + idx) * D;
+  float* o = centres + ((size_t)prob * C + c) * D;
+  for (int d = threadIdx.x; d < D; d += blockDim.x) o[d] = to_f(x[d]);
+}
+
+__global__ void k_centre_norms(const float* __restrict__ centres, int total, int D, float* __restrict__ cnorm) {
+  const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (w >= total) return;
+  const float* c = centres + (size_t)w * D;
+  float s = 0.f;
+  for (int d = lane; d < D; d += 32) s = fmaf(c[d], c[d], s);
+  s = warp_sum(s);
+  if (lane == 0) cnorm[w] = s;
+}
+
+// Assignment: argmin_c |c|^2 - 2 x.c, fp32 FFMA, 128 points x 64 centres per tile, 8x4 per thread.
+constexpr int kAsgRows = 128, kAsgCols = 64, kAsgThreads = 256;
+
+template <class T, int D>
+__global__ void __launch_bounds__(kAsgThreads)
+k_assign(const T* __restrict__ X, int N, int C, const float* __restrict__ centres,
+         const float* __restrict__ cnorm, int32_t* __restrict__ assign) {
+  constexpr int LD = D + 4;
+  extern __shared__ float smf[];
+  float* Xs = smf;                       // [128][LD]
+  float* Cs = Xs + kAsgRows * LD;        // [64][LD]
+  float* cn = Cs + kAsgCols * LD;        // [64]
+  const int prob = blockIdx.y, row0 = blockIdx.x * kAsgRows;
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const T* Xp = X + (size_t)prob * N * D;
+  const float* Cp = centres + (size_t)prob * C * D;
+  const float* cnp = cnorm + (size_t)prob * C;
+  for (int e = tid; e < kAsgRows * (D / 4); e += kAsgThreads) {
+    int r = e / (D / 4), q = e % (D / 4);
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (row0 + r < N) v = ld4(Xp + (size_t)(row0 + r) * D + q * 4);
+    st4(Xs + r * LD + q * 4, v);
+  }
+  float best[8]; int bidx[8];
+#pragma unroll
+  for (int r = 0; r < 8; ++r) { best[r] = INFINITY; bidx[r] = 0x7fffffff; }
+  for (int c0 = 0; c0 < C; c0 += kAsgCols) {
+    __syncthreads();
+    for (int e = tid; e < kAsgCols * (D / 4); e += kAsgThreads) {
+      int r = e / (D / 4), q = e % (D / 4);
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (c0 + r < C) v = ld4(Cp + (size_t)(c0 + r) * D + q * 4);
+      st4(Cs + r * LD + q * 4, v);
+    }
+    if (tid < kAsgCols) cn[tid] = (c0 + tid < C) ? cnp[c0 + tid] : INFINITY;
+    __syncthreads();
+    float acc[8][4];
+#pragma unroll
+    for (int r = 0; r < 8; ++r)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) acc[r][k] = 0.f;
+#pragma unroll 4
+    for (int d = 0; d < D; d += 4) {
+      float4 cv[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) cv[k] = ld4(Cs + (tx * 4 + k) * LD + d);
+#pragma unroll
+      for (int r = 0; r < 8; ++r) {
+        float4 xv = ld4(Xs + (ty * 8 + r) * LD + d);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          acc[r][k] = fmaf(xv.x, cv[k].x, acc[r][k]);
+          acc[r][k] = fmaf(xv.y, cv[k].y, acc[r][k]);
+          acc[r][k] = fmaf(xv.z, cv[k].z, acc[r][k]);
+          acc[r][k] = fmaf(xv.w, cv[k].w, acc[r][k]);
+        }
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < 8; ++r)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        float dist = fmaf(-2.f, acc[r][k], cn[tx * 4 + k]);
+        int c = c0 + tx * 4 + k;
+        if (dist < best[r]) { best[r] = dist; bidx[r] = c; }   // ascending c: ties keep the lower
+      }
+  }
+#pragma unroll
+  for (int r = 0; r < 8; ++r) {
+    float b = best[r]; int i = bidx[r];
+#pragma unroll
+    for (int o = 8; o > 0; o >>= 1) {
+      float ob = __shfl_xor_sync(0xffffffffu, b, o);
+      int oi = __shfl_xor_sync(0xffffffffu, i, o);
+      if (ob < b || (ob == b && oi < i)) { b = ob; i = oi; }
+    }
+    int row = row0 + ty * 8 + r;
+    if (tx == 0 && row < N) assign[(size_t)prob * N + row] = i;
+  }
+}
+
+// Centre update: mean of the members, summed in bucket order with a fixed reduction tree, so
+// the result does not depend on scheduling.  An empty cluster keeps its centre.
+template <class T, int D>
+__global__ void __launch_bounds__(128)
+k_update(const T* __restrict__ X, int N, int C, int S, int kind, const int32_t* __restrict__ off,
+         const int32_t* __restrict__ perm, float* __restrict__ centres, float* __restrict__ cnorm) {
+  constexpr int LPR = D / 4;            // lanes per row
+  constexpr int RPW = 32 / LPR;         // rows per warp step
+  constexpr int SLOTS = 4 * RPW;
+  __shared__ float4 part[SLOTS][LPR];
+  const int c = blockIdx.x, prob = blockIdx.y;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int sub = lane / LPR, q = lane % LPR;
+  const int slot = warp * RPW + sub;
+  const T* Xp = X + (size_t)prob * N * D;
+  const int32_t* o = off + (size_t)prob * (C * S + 1);
+  const int32_t* pm = perm + (size_t)prob * N;
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  int count = 0;
+  const int nranges = kind == 0 ? S : 1;
+  for (int r = 0; r < nranges; ++r) {
+    int p0 = kind == 0 ? o[r * C + c] : o[c * S];
+    int p1 = kind == 0 ? o[r * C + c + 1] : o[(c + 1) * S];
+    count += p1 - p0;
+    for (int p = p0 + slot; p < p1; p += SLOTS) {
+      float4 v = ld4(Xp + (size_t)pm[p] * D + q * 4);
+      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    }
+  }
+  part[slot][q] = s;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
+    float* dst = centres + ((size_t)prob * C + c) * D;
+    if (lane < LPR) {
+      for (int k = 0; k < SLOTS; ++k) { float4 v = part[k][lane]; tot.x += v.x; tot.y += v.y; tot.z += v.z; tot.w += v.w; }
+      if (count > 0) {
+        float inv = 1.f / (float)count;
+        tot.x *= inv; tot.y *= inv; tot.z *= inv; tot.w *= inv;
+        st4(dst + lane * 4, tot);
+      } else {
+        tot = ld4(dst + lane * 4);
+      }
+    }
+    float n2 = tot.x * tot.x + tot.y * tot.y + tot.z * tot.z + tot.w * tot.w;
+    n2 = warp_sum(n2);
+    if (lane == 0) cnorm[(size_t)prob * C + c] = n2;
+  }
+}
+
+template <class T, int D>
+static int lloyd_t(const Dims& d, const T* X, int problems, int C, int kind, const int32_t* init_idx,
+                   int init_mode, uint64_t seed, int T_iters, int32_t* assign, float* centres, void* ws,
+                   cudaStream_t st) {
+  Arena ar(ws);
+  float* cnorm = ar.take<float>((size_t)problems * C);
+  int32_t* off = ar.take<int32_t>((size_t)problems * (C * d.S + 1));
+  int32_t* perm = ar.take<int32_t>((size_t)problems * d.N);
+  int32_t* scratch = ar.take<int32_t>((size_t)problems * sort_ws_elems(d.N, C * d.S));
+  if (init_mode != MUSE_INIT_CENTRES) {
+    k_init_centres<T><<<dim3(C, problems), 32, 0, st>>>(X, d.N, D, C, init_idx, init_mode, seed, kind, centres);
+    MUSE_LAUNCH_OK();
+  }
+  const int total = problems * C;
+  k_centre_norms<<<cdiv(total * 32, 256), 256, 0, st>>>(centres, total, D, cnorm);
+  MUSE_LAUNCH_OK();
+  const size_t smem = (size_t)((kAsgRows + kAsgCols) * (D + 4) + kAsgCols) * sizeof(float);
+  MUSE_CUDA_OK(cudaFuncSetAttribute(k_assign<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  for (int it = 0; it <= T_iters; ++it) {
+    k_assign<T, D><<<dim3(cdiv(d.N, kAsgRows), problems), kAsgThreads, smem, st>>>(X, d.N, C, centres, cnorm, assign);
+    MUSE_LAUNCH_OK();
+    if (it == T_iters) break;
+    int rc = bucket_sort(0, assign, problems, d.N, C, d.S, d.Bs, kind, off, perm, scratch, st);
+    if (rc != MUSE_OK) return rc;
+    k_update<T, D><<<dim3(C, problems), 128, 0, st>>>(X, d.N, C, d.S, kind, off, perm, centres, cnorm);
+    MUSE_LAUNCH_OK();
+  }
+  return MUSE_OK;
+}
+
+size_t lloyd_ws_bytes(const Dims& d, int problems, int C, int) {
+  Arena ar(nullptr);
+  ar.take<float>((size_t)problems * C);
+  ar.take<int32_t>((size_t)problems * (C * d.S + 1));
+  ar.take<int32_t>((size_t)problems * d.N);
+  ar.take<int32_t>((size_t)problems * sort_ws_elems(d.N, C * d.S));
+  return ar.used;
+}
+
+int lloyd(const Dims& d, int dtype, const void* X, int problems, int C, int kind, const int32_t* init_idx,
+          int init_mode, uint64_t seed, int T, int32_t* assign, float* centres, void* ws, cudaStream_t st) {
+  if (dtype == MUSE_F32) {
+    if (d.D == 64) return lloyd_t<float, 64>(d, (const float*)X, problems, C, kind, init_idx, init_mode, seed, T, assign, centres, ws, st);
+    return lloyd_t<float, 128>(d, (const float*)X, problems, C, kind, init_idx, init_mode, seed, T, assign, centres, ws, st);
+  }
+  if (d.D == 64) return lloyd_t<__nv_bfloat16, 64>(d, (const __nv_bfloat16*)X, problems, C, kind, init_idx, init_mode, seed, T, assign, centres, ws, st);
+  return lloyd_t<__nv_bfloat16, 128>(d, (const __nv_bfloat16*)X, problems, C, kind, init_idx, init_mode, seed, T, assign, centres, ws, st);
+}
+
+}  // namespace muse

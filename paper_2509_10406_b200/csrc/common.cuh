@@ -1,0 +1,118 @@
+// Shared declarations of the MuSe CUDA library (internal; the public C ABI is include/muse.h).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include <math.h>
+#include "../../include/muse.h"
+
+namespace muse {
+
+constexpr int kMaxHeads = 128;
+constexpr int kMaxM = 64;
+constexpr int kMaxC = 4096;
+
+struct HeadMap { int16_t g[kMaxHeads]; };
+
+// Resolved problem description passed by value to kernels.
+struct Dims {
+  int B, Hq, Hkv, N, D, Cq, Ck, m;
+  int S;        // spatial blocks (1 when non-causal)
+  int SB;       // stored summary planes: S-1 (causal) or 1
+  int Bs;       // block size N / S
+  int causal, sel_mode, agg_grad;
+  float sigma;
+  HeadMap hm;
+};
+
+#define MUSE_CUDA_OK(expr) do { cudaError_t e_ = (expr); if (e_ != cudaSuccess) return MUSE_ERR_CUDA; } while (0)
+#define MUSE_LAUNCH_OK() do { if (cudaPeekAtLastError() != cudaSuccess) { cudaGetLastError(); return MUSE_ERR_CUDA; } } while (0)
+
+// Bump allocator over the caller's workspace (256-byte granularity); with base == nullptr it
+// only measures.
+struct Arena {
+  char* base; size_t used;
+  explicit Arena(void* b) : base(static_cast<char*>(b)), used(0) {}
+  template <class T> T* take(size_t count) {
+    size_t bytes = (count * sizeof(T) + 255) & ~size_t(255);
+    T* p = base ? reinterpret_cast<T*>(base + used) : nullptr;
+    used += bytes;
+    return p;
+  }
+};
+
+__host__ __device__ inline int cdiv(int a, int b) { return (a + b - 1) / b; }
+
+// ---- element access -----------------------------------------------------------------------
+__device__ __forceinline__ float to_f(float x) { return x; }
+__device__ __forceinline__ float to_f(__nv_bfloat16 x) { return __bfloat162float(x); }
+template <class T> __device__ __forceinline__ T from_f(float x);
+template <> __device__ __forceinline__ float from_f<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// Load 4 consecutive elements (16-byte aligned for float, 8-byte for bf16) as floats.
+__device__ __forceinline__ float4 ld4(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 ld4(const __nv_bfloat16* p) {
+  uint2 u = *reinterpret_cast<const uint2*>(p);
+  float4 r;
+  r.x = __uint_as_float(u.x << 16); r.y = __uint_as_float(u.x & 0xffff0000u);
+  r.z = __uint_as_float(u.y << 16); r.w = __uint_as_float(u.y & 0xffff0000u);
+  return r;
+}
+__device__ __forceinline__ void st4(float* p, float4 v) { *reinterpret_cast<float4*>(p) = v; }
+__device__ __forceinline__ void st4(__nv_bfloat16* p, float4 v) {
+  __nv_bfloat162 a = __floats2bfloat162_rn(v.x, v.y), b = __floats2bfloat162_rn(v.z, v.w);
+  uint2 u; u.x = *reinterpret_cast<uint32_t*>(&a); u.y = *reinterpret_cast<uint32_t*>(&b);
+  *reinterpret_cast<uint2*>(p) = u;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// ---- stage launchers (each enqueues on `st`, returns MUSE_OK or MUSE_ERR_CUDA) ---------------
+// clustering side: kind 0 = queries (key = block*C + cluster), kind 1 = keys (key = cluster*S + block)
+size_t sort_ws_elems(int N, int nkeys);   // int32 scratch elements per problem for bucket_sort
+int bucket_sort(int dtype_unused, const int32_t* assign, int problems, int N, int C, int S, int Bs,
+                int kind, int32_t* off, int32_t* perm, int32_t* scratch, cudaStream_t st);
+
+int lloyd(const Dims& d, int dtype, const void* X, int problems, int C, int kind,
+          const int32_t* init_idx, int init_mode, uint64_t seed, int T,
+          int32_t* assign, float* centres, void* ws, cudaStream_t st);
+size_t lloyd_ws_bytes(const Dims& d, int problems, int C, int kind);
+
+int summarize(const Dims& d, int dtype, const void* K, const void* V, const int32_t* assign_k,
+              const float* qbar, int32_t* off_k, int32_t* perm_k, void* summaries, void* ws,
+              cudaStream_t st);
+size_t summarize_ws_bytes(const Dims& d);
+
+struct SummLayout { size_t mu, kappa, nu, Kp, Vp, total; };
+SummLayout summ_layout(const Dims& d, int dtype);
+
+int attn_fwd(const Dims& d, int dtype, const void* Q, const void* K, const void* V,
+             const int32_t* assign_q, const float* qbar, const int32_t* off_k, const int32_t* perm_k,
+             const void* summaries, const int32_t* sel_in, void* O, float* LSE, int32_t* sel_out,
+             void* ws, cudaStream_t st);
+size_t attn_fwd_ws_bytes(const Dims& d, int dtype);
+
+int attn_bwd(const Dims& d, int dtype, const void* Q, const void* K, const void* V, const void* O,
+             const float* LSE, const void* dO, const int32_t* assign_q, const float* qbar,
+             const int32_t* off_k, const int32_t* perm_k, const void* summaries, const int32_t* sel,
+             void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
+size_t attn_bwd_ws_bytes(const Dims& d, int dtype);
+
+// retrieval inverse index, shared by forward and backward: groups the (query, slot) pairs by
+// (query block - 1, key cluster).  pair id = t * m + slot.
+struct RetIndex { int32_t* goff; int32_t* pairs; int32_t* cursor; };
+size_t ret_index_elems(const Dims& d);     // int32 elements per query head
+int build_ret_index(const Dims& d, const int32_t* sel, int32_t* scratch, RetIndex* out, cudaStream_t st);
+
+}  // namespace muse

@@ -1,0 +1,194 @@
+// Summaries stage: bucket keys by (cluster, block), then build the exclusive causal
+// accumulation of the exponentially tilted per-block summaries (Section "Summary Computation
+// and Causal Accumulation", Eq. 3-5; Algorithm 1 "Causal accumulation along spatial axis").
+#include "common.cuh"
+
+namespace muse {
+
+SummLayout summ_layout(const Dims& d, int dtype) {
+  const size_t es = dtype == MUSE_F32 ? 4 : 2;
+  const size_t ent = (size_t)d.B * d.Hq * d.SB * d.Cq * d.Ck;
+  auto up = [](size_t x) { return (x + 255) & ~size_t(255); };
+  SummLayout L;
+  L.mu = 0;
+  L.kappa = up(L.mu + ent * sizeof(float));
+  L.nu = up(L.kappa + ent * d.D * sizeof(float));
+  L.Kp = up(L.nu + ent * d.D * sizeof(float));
+  L.Vp = up(L.Kp + (size_t)d.B * d.Hkv * d.N * d.D * es);
+  L.total = up(L.Vp + (size_t)d.B * d.Hkv * d.N * d.D * es);
+  return L;
+}
+
+// out[p] = in[perm[p]] for whole rows of D elements (16 bytes per thread).
+template <class T>
+__global__ void k_gather_rows(const T* __restrict__ in, const int32_t* __restrict__ perm, int N, int D,
+                              T* __restrict__ out) {
+  const int vpr = D * (int)sizeof(T) / 16;           // 16-byte vectors per row
+  const int prob = blockIdx.y;
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= (long long)N * vpr) return;
+  const int p = (int)(e / vpr), v = (int)(e % vpr);
+  const uint4* src = reinterpret_cast<const uint4*>(in + ((size_t)prob * N + perm[(size_t)prob * N + p]) * D);
+  uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)prob * N + p) * D);
+  dst[v] = src[v];
+}
+
+// One CTA = (key cluster j, tile of 64 query clusters, query head).  It walks the cluster's
+// buckets in block order, keeping for each query centroid i a running (max, mass, weighted
+// sums of [k|v]) exactly like an online softmax, and emits a normalised snapshot after each
+// bucket: the snapshot after bucket b is the accumulated summary seen by queries of block b+1.
+constexpr int kSumI = 64, kSumKC = 16, kSumThreads = 256;
+
+template <class T, int D>
+__global__ void __launch_bounds__(kSumThreads)
+k_summarize(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const int32_t* __restrict__ off_k,
+            const float* __restrict__ qbar, float* __restrict__ mu, float* __restrict__ kappa,
+            float* __restrict__ nu) {
+  constexpr int LDQ = D + 4, LDKV = 2 * D + 4, LDL = kSumKC + 1, NV = 2 * D / 32;
+  extern __shared__ float smf[];
+  float* qb = smf;                         // [64][LDQ]  sigma * qbar tile
+  float* kv = qb + kSumI * LDQ;            // [KC][LDKV] rows [k | v]
+  float* Ls = kv + kSumKC * LDKV;          // [64][LDL]  tilt logits
+  const int j = blockIdx.x, i0 = blockIdx.y * kSumI, pq = blockIdx.z;
+  const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
+  const int tid = threadIdx.x;
+  const float* qsrc = qbar + (size_t)pq * dm.Cq * D;
+  for (int e = tid; e < kSumI * (D / 4); e += kSumThreads) {
+    int r = e / (D / 4), q = e % (D / 4);
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (i0 + r < dm.Cq) v = ld4(qsrc + (size_t)(i0 + r) * D + q * 4);
+    v.x *= dm.sigma; v.y *= dm.sigma; v.z *= dm.sigma; v.w *= dm.sigma;
+    st4(qb + r * LDQ + q * 4, v);
+  }
+  const int32_t* off = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
+  const T* Kb = Kp + (size_t)pk * dm.N * D;
+  const T* Vb = Vp + (size_t)pk * dm.N * D;
+  const int ip = tid >> 3, sl = tid & 7;           // phase 2: i pair, dim slice
+  const int li = tid >> 2, ug = tid & 3;           // phase 1: i, group of 4 keys
+  float acc[2][NV][4];
+  float M[2] = {-INFINITY, -INFINITY}, s[2] = {0.f, 0.f};
+#pragma unroll
+  for (int a = 0; a < 2; ++a)
+#pragma unroll
+    for (int k = 0; k < NV; ++k)
+#pragma unroll
+      for (int c = 0; c < 4; ++c) acc[a][k][c] = 0.f;
+
+  for (int b = 0; b < dm.SB; ++b) {
+    const int p0 = off[b], p1 = off[b + 1];
+    for (int c0 = p0; c0 < p1; c0 += kSumKC) {
+      const int n = min(kSumKC, p1 - c0);
+      __syncthreads();
+      for (int e = tid; e < n * (2 * D / 4); e += kSumThreads) {
+        int r = e / (2 * D / 4), q = e % (2 * D / 4);
+        float4 v = q < D / 4 ? ld4(Kb + (size_t)(c0 + r) * D + q * 4)
+                             : ld4(Vb + (size_t)(c0 + r) * D + (q - D / 4) * 4);
+        st4(kv + r * LDKV + q * 4, v);
+      }
+      __syncthreads();
+      {
+        float dot[4] = {0.f, 0.f, 0.f, 0.f};
+        if (ug * 4 < n) {
+#pragma unroll 4
+          for (int dd = 0; dd < D; dd += 4) {
+            float4 qv = ld4(qb + li * LDQ + dd);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              float4 kk = ld4(kv + (ug * 4 + u) * LDKV + dd);   // rows >= n hold stale finite data; unused
+              dot[u] = fmaf(qv.x, kk.x, dot[u]); dot[u] = fmaf(qv.y, kk.y, dot[u]);
+              dot[u] = fmaf(qv.z, kk.z, dot[u]); dot[u] = fmaf(qv.w, kk.w, dot[u]);
+            }
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) Ls[li * LDL + ug * 4 + u] = dot[u];
+      }
+      __syncthreads();
+#pragma unroll
+      for (int a = 0; a < 2; ++a) {
+        const float* Lr = Ls + (ip * 2 + a) * LDL;
+        float cm = -INFINITY;
+        for (int u = 0; u < n; ++u) cm = fmaxf(cm, Lr[u]);
+        const float Mn = fmaxf(M[a], cm);
+        const float sc = expf(M[a] - Mn);            // exp(-inf) = 0 on the first keys
+        M[a] = Mn; s[a] *= sc;
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) acc[a][k][c] *= sc;
+        for (int u = 0; u < n; ++u) {
+          const float w = expf(Lr[u] - Mn);
+          s[a] += w;
+#pragma unroll
+          for (int k = 0; k < NV; ++k) {
+            float4 x = ld4(kv + u * LDKV + sl * 4 + 32 * k);
+            acc[a][k][0] = fmaf(w, x.x, acc[a][k][0]); acc[a][k][1] = fmaf(w, x.y, acc[a][k][1]);
+            acc[a][k][2] = fmaf(w, x.z, acc[a][k][2]); acc[a][k][3] = fmaf(w, x.w, acc[a][k][3]);
+          }
+        }
+      }
+    }
+    // snapshot -> plane b
+#pragma unroll
+    for (int a = 0; a < 2; ++a) {
+      const int i = i0 + ip * 2 + a;
+      if (i >= dm.Cq) continue;
+      const size_t ent = (((size_t)pq * dm.SB + b) * dm.Cq + i) * dm.Ck + j;
+      const bool some = s[a] > 0.f;
+      const float inv = some ? 1.f / s[a] : 0.f;
+      if (sl == 0) mu[ent] = some ? M[a] + logf(s[a]) : -INFINITY;
+#pragma unroll
+      for (int k = 0; k < NV; ++k) {
+        const int c4 = sl * 4 + 32 * k;
+        float4 v = make_float4(acc[a][k][0] * inv, acc[a][k][1] * inv, acc[a][k][2] * inv, acc[a][k][3] * inv);
+        if (c4 < D) st4(kappa + ent * D + c4, v);
+        else st4(nu + ent * D + (c4 - D), v);
+      }
+    }
+  }
+}
+
+template <class T, int D>
+static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const int32_t* assign_k,
+                       const float* qbar, int32_t* off_k, int32_t* perm_k, void* summaries, void* ws,
+                       cudaStream_t st) {
+  const int pk = d.B * d.Hkv;
+  int rc = bucket_sort(0, assign_k, pk, d.N, d.Ck, d.S, d.Bs, 1, off_k, perm_k, (int32_t*)ws, st);
+  if (rc != MUSE_OK) return rc;
+  SummLayout L = summ_layout(d, dtype);
+  char* base = (char*)summaries;
+  T* Kp = (T*)(base + L.Kp); T* Vp = (T*)(base + L.Vp);
+  const int vpr = D * (int)sizeof(T) / 16;
+  dim3 gg(cdiv(d.N * vpr, 256), pk);
+  k_gather_rows<T><<<gg, 256, 0, st>>>(K, perm_k, d.N, D, Kp);
+  MUSE_LAUNCH_OK();
+  k_gather_rows<T><<<gg, 256, 0, st>>>(V, perm_k, d.N, D, Vp);
+  MUSE_LAUNCH_OK();
+  if (d.SB == 0) return MUSE_OK;
+  const size_t smem = (size_t)(kSumI * (D + 4) + kSumKC * (2 * D + 4) + kSumI * (kSumKC + 1)) * sizeof(float);
+  MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  dim3 grid(d.Ck, cdiv(d.Cq, kSumI), d.B * d.Hq);
+  k_summarize<T, D><<<grid, kSumThreads, smem, st>>>(d, Kp, Vp, off_k, qbar, (float*)(base + L.mu),
+                                                    (float*)(base + L.kappa), (float*)(base + L.nu));
+  MUSE_LAUNCH_OK();
+  return MUSE_OK;
+}
+
+size_t summarize_ws_bytes(const Dims& d) {
+  Arena ar(nullptr);
+  ar.take<int32_t>((size_t)d.B * d.Hkv * sort_ws_elems(d.N, d.Ck * d.S));
+  return ar.used;
+}
+
+int summarize(const Dims& d, int dtype, const void* K, const void* V, const int32_t* assign_k,
+              const float* qbar, int32_t* off_k, int32_t* perm_k, void* summaries, void* ws, cudaStream_t st) {
+  if (dtype == MUSE_F32) {
+    if (d.D == 64) return summarize_t<float, 64>(d, dtype, (const float*)K, (const float*)V, assign_k, qbar, off_k, perm_k, summaries, ws, st);
+    return summarize_t<float, 128>(d, dtype, (const float*)K, (const float*)V, assign_k, qbar, off_k, perm_k, summaries, ws, st);
+  }
+  typedef __nv_bfloat16 bf;
+  if (d.D == 64) return summarize_t<bf, 64>(d, dtype, (const bf*)K, (const bf*)V, assign_k, qbar, off_k, perm_k, summaries, ws, st);
+  return summarize_t<bf, 128>(d, dtype, (const bf*)K, (const bf*)V, assign_k, qbar, off_k, perm_k, summaries, ws, st);
+}
+
+}  // namespace muse

@@ -1,0 +1,124 @@
+"""GPU parity: summaries and forward attention against the fp64 oracle, teacher-forced
+(identical assignments and query centroids on both sides).  Tolerance: max-abs error
+relative to the oracle tensor's max-abs <= 1e-4 in fp32 mode, 2e-2 in bf16 mode."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import muse_oracle as orc
+from paper_2509_10406_b200 import workloads as wl
+from tests.gpu_util import Case, to_dev, to_np, tol, rel_err
+from tests.test_gpu_cluster import CASES
+
+pytestmark = pytest.mark.gpu
+
+EDGE = {
+    "m0": CASES["gqa_bf16"].with_(B=1, Hq=2, Hkv=1, m=0),
+    "one_block": CASES["tiny"].with_(S=1),
+    "one_qcluster": CASES["tiny"].with_(Cq=1, N=512),
+    "tiny_blocks": CASES["tiny"].with_(N=64, Cq=2, Ck=8, m=8, components=4),
+    "ragged_f32_d128": CASES["d128"].with_(dtype="f32", N=1000, Hq=1, Cq=8, Ck=24, m=3),
+}
+
+
+def _mb():
+    from paper_2509_10406_b200 import binding as mb
+    return mb
+
+
+def _run_summaries(mb, c, p, buf, K, V):
+    mb.muse_summarize(p, K, V, to_dev(c.a_k, "i"), to_dev(c.qbar32, "f32"), buf.off_k, buf.perm_k, buf.summaries, buf.ws)
+
+
+def _prep(w, gain, **pk):
+    mb = _mb()
+    c = Case(w, gain=gain)
+    c.qbar32 = c.qbar.astype(np.float32)
+    p = c.params(**pk)
+    buf = mb.MuseBuffers(p, backward=True)
+    return mb, c, p, buf
+
+
+@pytest.mark.parametrize("name", list(CASES))
+@pytest.mark.parametrize("gain", [1.0, 128.0])
+def test_summaries_match_oracle(name, gain):
+    mb, c, p, buf = _prep(CASES[name], gain)
+    w = c.w
+    Q, K, V, _ = c.dev()
+    _run_summaries(mb, c, p, buf, K, V)
+    torch.cuda.synchronize()
+    mu, ka, nu = (to_np(x) for x in buf.summary_planes())
+    for b in range(w.B):
+        for h in range(w.Hq):
+            g = c.hm[h]
+            muh, kah, nuh = orc.accumulated_summaries(c.K[b, g], c.V[b, g], c.a_k[b, g], c.qbar32[b, h].astype(np.float64),
+                                                      c.sigma, w.S, w.Ck)
+            e_mu, g_mu = muh[1:], mu[b, h]
+            assert np.array_equal(np.isfinite(e_mu), np.isfinite(g_mu))
+            fin = np.isfinite(e_mu)
+            assert np.abs(e_mu[fin] - g_mu[fin]).max() <= 1e-4 * max(1.0, np.abs(e_mu[fin]).max())
+            assert rel_err(ka[b, h], kah[1:]) <= 1e-4
+            assert rel_err(nu[b, h], nuh[1:]) <= 1e-4
+
+
+def _forward_parity(w, gain, sel_mode=0, causal=True):
+    mb, c, p, buf = _prep(w, gain, sel_mode=sel_mode, causal=causal)
+    Q, K, V, _ = c.dev()
+    _run_summaries(mb, c, p, buf, K, V)
+    kw = dict(sigma=c.sigma, S=w.S, Ck=w.Ck, m=w.m, sel_mode=sel_mode, causal=causal)
+    t = tol(w.dtype)
+    # free selection on the GPU
+    mb.muse_attn_fwd(p, Q, K, V, to_dev(c.a_q, "i"), to_dev(c.qbar32, "f32"), buf.off_k, buf.perm_k, buf.summaries,
+                     None, buf.O, buf.LSE, buf.sel, buf.ws)
+    torch.cuda.synchronize()
+    O_free, L_free, sel_gpu = to_np(buf.O), to_np(buf.LSE), to_np(buf.sel)[..., :w.m]
+    stats = dict(sel_rows_differ=0, rows=0, err_forced_gpu_sel=0.0, err_forced_orc_sel=0.0)
+    sel_orc = np.full((w.B, w.Hq, w.N, max(w.m, 1)), -1, np.int32)
+    for b in range(w.B):
+        for h in range(w.Hq):
+            g = c.hm[h]
+            args = (c.Q[b, h], c.K[b, g], c.V[b, g], c.a_q[b, h], c.a_k[b, g], c.qbar32[b, h].astype(np.float64))
+            f = orc.forward(*args, **kw)
+            sel_orc[b, h, :, :w.m] = f["sel"]
+            # selections: equal as sets except where the oracle's margin is below tolerance
+            same = np.array([set(x) == set(y) for x, y in zip(f["sel"].tolist(), sel_gpu[b, h].tolist())])
+            assert np.all(f["sel_gap"][~same] < t), ("selection differs away from a near-tie", f["sel_gap"][~same].max())
+            stats["sel_rows_differ"] += int((~same).sum()); stats["rows"] += w.N
+            # outputs: oracle forced to the GPU's selections
+            ff = orc.forward(*args, sel=sel_gpu[b, h], summ=f["summ"], **kw)
+            e = max(rel_err(O_free[b, h], ff["O"]), float(np.abs(L_free[b, h] - ff["LSE"]).max() / max(1.0, np.abs(ff["LSE"]).max())))
+            stats["err_forced_gpu_sel"] = max(stats["err_forced_gpu_sel"], e)
+    assert stats["err_forced_gpu_sel"] <= t, stats
+    # GPU forced to the oracle's selections
+    mb.muse_attn_fwd(p, Q, K, V, to_dev(c.a_q, "i"), to_dev(c.qbar32, "f32"), buf.off_k, buf.perm_k, buf.summaries,
+                     to_dev(sel_orc, "i"), buf.O, buf.LSE, buf.sel, buf.ws)
+    torch.cuda.synchronize()
+    O_f = to_np(buf.O)
+    for b in range(w.B):
+        for h in range(w.Hq):
+            g = c.hm[h]
+            f = orc.forward(c.Q[b, h], c.K[b, g], c.V[b, g], c.a_q[b, h], c.a_k[b, g], c.qbar32[b, h].astype(np.float64),
+                            sel=sel_orc[b, h, :, :w.m], **kw)
+            stats["err_forced_orc_sel"] = max(stats["err_forced_orc_sel"], rel_err(O_f[b, h], f["O"]))
+    print(w.name, gain, stats)
+    assert stats["err_forced_orc_sel"] <= t, stats
+    assert stats["sel_rows_differ"] <= 0.02 * stats["rows"] + 2
+
+
+@pytest.mark.parametrize("name", list(CASES))
+@pytest.mark.parametrize("gain", [1.0, 128.0])
+def test_forward_matches_oracle(name, gain):
+    _forward_parity(CASES[name], gain)
+
+
+@pytest.mark.parametrize("name", list(EDGE))
+def test_forward_edge_cases(name):
+    _forward_parity(EDGE[name], 128.0)
+
+
+def test_forward_per_query_cluster_selection():
+    _forward_parity(CASES["gqa_bf16"], 128.0, sel_mode=1)
+
+
+def test_forward_noncausal():
+    _forward_parity(CASES["tiny"], 128.0, causal=False)
