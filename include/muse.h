@@ -142,6 +142,15 @@ MUSE_API int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K,
                   const int32_t* sel, void* dQ, void* dK, void* dV,
                   void* ws, size_t ws_bytes, cudaStream_t stream);
 
+/* Per-kernel timing for benchmarks (no counterpart in the paper).  muse_profile(1) clears the
+ * record and makes every later library call record CUDA events on its stream around each
+ * kernel launch (events are created on demand and reused); muse_profile(0) stops recording.
+ * muse_profile_report waits for the last recorded event, then writes one text line per kernel
+ * name, "name launches total_ms", into buf (HOST, cap bytes) and returns the byte count, or a
+ * negative MUSE_ERR_* code.  Not thread-safe with respect to concurrent library calls. */
+MUSE_API int muse_profile(int enable);
+MUSE_API long muse_profile_report(char* buf, size_t cap);
+
 /* Human-readable text for a return code (static storage). */
 MUSE_API const char* muse_strerror(int code);
 

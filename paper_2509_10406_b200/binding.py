@@ -21,7 +21,7 @@ MUSE_SEL_PER_QUERY, MUSE_SEL_PER_QCLUSTER = 0, 1
 MUSE_INIT_INDICES, MUSE_INIT_STRIDED, MUSE_INIT_CENTRES = 0, 1, 2
 
 EXPORTS = ("muse_workspace_bytes", "muse_summaries_layout", "muse_cluster", "muse_summarize",
-           "muse_attn_fwd", "muse_attn_bwd", "muse_strerror")
+           "muse_attn_fwd", "muse_attn_bwd", "muse_profile", "muse_profile_report", "muse_strerror")
 
 
 class MuseParams(ctypes.Structure):
@@ -83,8 +83,11 @@ def lib() -> ctypes.CDLL:
         L.muse_attn_fwd.argtypes = [pp, vp, vp, vp, i32p, f32p, i32p, i32p, vp, i32p, vp, f32p, i32p, vp, sz, vp]
         L.muse_attn_bwd.argtypes = [pp, vp, vp, vp, vp, f32p, vp, i32p, f32p, i32p, i32p, vp, i32p, vp, vp, vp,
                                     vp, sz, vp]
+        L.muse_profile.argtypes = [ctypes.c_int]
+        L.muse_profile_report.argtypes = [ctypes.c_char_p, sz]
         for name in EXPORTS[:-1]:
             getattr(L, name).restype = ctypes.c_int
+        L.muse_profile_report.restype = ctypes.c_long
         _lib = L
     return _lib
 
@@ -114,6 +117,23 @@ def muse_workspace_bytes(p: MuseParams):
     out = (ctypes.c_size_t * 5)()
     _check(lib().muse_workspace_bytes(ctypes.byref(p), out), "muse_workspace_bytes")
     return tuple(int(x) for x in out)
+
+
+def muse_profile(enable: bool) -> None:
+    _check(lib().muse_profile(int(enable)), "muse_profile")
+
+
+def muse_profile_report() -> dict:
+    """{kernel name: (launches, total ms)} since muse_profile(True)."""
+    buf = ctypes.create_string_buffer(1 << 16)
+    n = lib().muse_profile_report(buf, len(buf))
+    if n < 0:
+        _check(int(n), "muse_profile_report")
+    out = {}
+    for line in buf.value.decode().splitlines():
+        name, launches, ms = line.split()
+        out[name] = (int(launches), float(ms))
+    return out
 
 
 def muse_summaries_layout(p: MuseParams):

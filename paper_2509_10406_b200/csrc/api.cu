@@ -103,6 +103,7 @@ int muse_cluster(const muse_params_t* p, const void* Q, const void* K, const int
     rc = lloyd(d, p->dtype, K, d.B * d.Hkv, d.Ck, 1, init_k, p->init_mode, p->seed, p->kmeans_iters, assign_k, kcent, ws, stream);
     if (rc != MUSE_OK) return rc;
   }
+  prof_mark(nullptr, stream);
   return MUSE_OK;
 }
 
@@ -117,7 +118,9 @@ int muse_summarize(const muse_params_t* p, const void* K, const void* V, const i
   size_t need[5];
   muse_workspace_bytes(p, need);
   if (ws_bytes < need[1]) return MUSE_ERR_WORKSPACE;
-  return summarize(d, p->dtype, K, V, assign_k, qbar, off_k, perm_k, summaries, ws, stream);
+  rc = summarize(d, p->dtype, K, V, assign_k, qbar, off_k, perm_k, summaries, ws, stream);
+  prof_mark(nullptr, stream);
+  return rc;
 }
 
 int muse_attn_fwd(const muse_params_t* p, const void* Q, const void* K, const void* V,
@@ -132,7 +135,9 @@ int muse_attn_fwd(const muse_params_t* p, const void* Q, const void* K, const vo
   size_t need[5];
   muse_workspace_bytes(p, need);
   if (ws_bytes < need[2]) return MUSE_ERR_WORKSPACE;
-  return attn_fwd(d, p->dtype, Q, K, V, assign_q, qbar, off_k, perm_k, summaries, sel_in, O, LSE, sel_out, ws, stream);
+  rc = attn_fwd(d, p->dtype, Q, K, V, assign_q, qbar, off_k, perm_k, summaries, sel_in, O, LSE, sel_out, ws, stream);
+  prof_mark(nullptr, stream);
+  return rc;
 }
 
 int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K, const void* V, const void* O,
@@ -149,7 +154,9 @@ int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K, const vo
   size_t need[5];
   muse_workspace_bytes(p, need);
   if (ws_bytes < need[3]) return MUSE_ERR_WORKSPACE;
-  return attn_bwd(d, p->dtype, Q, K, V, O, LSE, dO, assign_q, qbar, off_k, perm_k, summaries, sel, dQ, dK, dV, ws, stream);
+  rc = attn_bwd(d, p->dtype, Q, K, V, O, LSE, dO, assign_q, qbar, off_k, perm_k, summaries, sel, dQ, dK, dV, ws, stream);
+  prof_mark(nullptr, stream);
+  return rc;
 }
 
 }  // extern "C"

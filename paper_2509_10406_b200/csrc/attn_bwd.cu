@@ -675,8 +675,10 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
   const float* nu = (const float*)(base + L.nu);
   const size_t nd = (size_t)pq * d.N * d.D * sizeof(float);
   const long long rows = (long long)pq * d.N;
+  prof_mark("k_delta", st);
   k_delta<T, D><<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(O, dO, rows, w.delta);
   MUSE_LAUNCH_OK();
+  prof_mark("memset", st);
   MUSE_CUDA_OK(cudaMemsetAsync(w.dK_perm, 0, nd, st));
   MUSE_CUDA_OK(cudaMemsetAsync(w.dV_perm, 0, nd, st));
   const size_t sm4 = 4 * tile_bytes<T, D>() + ptile_bytes();
@@ -684,11 +686,14 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_local_bwd_dkdv<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm4));
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_local_bwd_dq<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm4));
     dim3 grid(d.S * cdiv(d.Bs, kTile), pq);
+    prof_mark("k_local_bwd_dkdv", st);
     k_local_bwd_dkdv<T, D><<<grid, kFlashThreads, sm4, st>>>(d, Q, K, V, dO, LSE, w.delta, w.dK_orig, w.dV_orig);
     MUSE_LAUNCH_OK();
+    prof_mark("k_local_bwd_dq", st);
     k_local_bwd_dq<T, D><<<grid, kFlashThreads, sm4, st>>>(d, Q, K, V, dO, LSE, w.delta, w.dQacc);
     MUSE_LAUNCH_OK();
   } else {
+    prof_mark("memset", st);
     MUSE_CUDA_OK(cudaMemsetAsync(w.dQacc, 0, nd, st));
   }
   int use_ret = 0;
@@ -700,6 +705,7 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
       rc = build_ret_index(d, sel, w.ret_scratch, &ri, st);
       if (rc != MUSE_OK) return rc;
       MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm4));
+      prof_mark("k_ret_bwd", st);
       k_ret_bwd<T, D><<<dim3(d.Ck, pq), kFlashThreads, sm4, st>>>(d, Q, dO, Kp, Vp, LSE, w.delta, off_k, ri.goff, ri.pairs,
                                                                 w.dq_part, w.dK_perm, w.dV_perm);
       MUSE_LAUNCH_OK();
@@ -707,17 +713,21 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
     }
     const size_t fsm = (size_t)(4 * kTile * (D + 4) + kTile * kLDP) * sizeof(float) + (size_t)kTile * cdiv(d.Ck, 32) * sizeof(uint32_t);
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fsm));
+    prof_mark("k_far_bwd", st);
     k_far_bwd<T, D><<<dim3(d.Cq, d.SB, pq), kFlashThreads, fsm, st>>>(d, Q, dO, qbar, LSE, w.delta, w.off_q, w.perm_q, sel, mu,
                                                                     kappa, nu, w.dQacc, w.dkappa, w.dnu, w.dS);
     MUSE_LAUNCH_OK();
     const size_t ssm = (size_t)(5 * kTile * (D + 4) + kTile * kLDP) * sizeof(float);
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
+    prof_mark("k_summ_bwd", st);
     k_summ_bwd<T, D><<<dim3(d.Ck, pq), kFlashThreads, ssm, st>>>(d, Kp, Vp, off_k, w.off_q, qbar, mu, w.dkappa, w.dnu, w.dS,
                                                                w.dK_perm, w.dV_perm);
     MUSE_LAUNCH_OK();
   }
+  prof_mark("k_final_dq", st);
   k_final_dq<T, D><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.dQacc, w.dq_part, sel, use_ret, dQ);
   MUSE_LAUNCH_OK();
+  prof_mark("k_final_dkv", st);
   k_final_dkv<T, D><<<dim3(cdiv(d.N * (D / 4), 256), pk), 256, 0, st>>>(d, perm_k, w.dK_orig, w.dV_orig, w.dK_perm, w.dV_perm,
                                                                        d.causal, dK, dV);
   MUSE_LAUNCH_OK();

@@ -56,12 +56,15 @@ int build_ret_index(const Dims& d, const int32_t* sel, int32_t* scratch, RetInde
   // note: cursor / goff are indexed with their natural strides (nkeys, nkeys + 1); the padded
   // region sizes above only reserve space
   if (d.m == 0 || nkeys == 0) return MUSE_OK;
+  prof_mark("memset", st);
   MUSE_CUDA_OK(cudaMemsetAsync(out->cursor, 0, (size_t)pq * nkeys * sizeof(int32_t), st));
   dim3 grid(cdiv((long long)d.N * d.m > 0 ? d.N * d.m : 1, 256), pq);
+  prof_mark("k_ret_count", st);
   k_ret_count<<<grid, 256, 0, st>>>(d, sel, out->cursor);
   MUSE_LAUNCH_OK();
   int rc = launch_scan(out->cursor, pq, nkeys, 1, out->goff, st);
   if (rc != MUSE_OK) return rc;
+  prof_mark("k_ret_fill", st);
   k_ret_fill<<<grid, 256, 0, st>>>(d, sel, out->cursor, out->pairs);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
@@ -508,9 +511,11 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
   // local attention
   if (d.causal) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_local_fwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fl_smem));
+    prof_mark("k_local_fwd", st);
     k_local_fwd<T, D><<<dim3(d.S * cdiv(d.Bs, kTile), pq), kFlashThreads, fl_smem, st>>>(d, Q, K, V, w.o_loc, w.lse_loc);
     MUSE_LAUNCH_OK();
   }
+  prof_mark("k_far_defaults", st);
   k_far_defaults<<<dim3(cdiv(d.N, 256), pq), 256, 0, st>>>(d, w.lse_far, sel);
   MUSE_LAUNCH_OK();
   if (d.SB > 0) {
@@ -518,6 +523,7 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
     if (rc != MUSE_OK) return rc;
     const size_t fs = far_smem(d.Ck, D);
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_fwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fs));
+    prof_mark("k_far_fwd", st);
     k_far_fwd<T, D><<<dim3(d.Cq, d.SB, pq), kFarThreads, fs, st>>>(
         d, Q, qbar, w.off_q, w.perm_q, (const float*)(base + L.mu), (const float*)(base + L.kappa),
         (const float*)(base + L.nu), sel_in, sel, w.o_far, w.lse_far);
@@ -527,10 +533,12 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
       rc = build_ret_index(d, sel, w.ret_scratch, &ri, st);
       if (rc != MUSE_OK) return rc;
       MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fl_smem));
+      prof_mark("k_ret_fwd", st);
       k_ret_fwd<T, D><<<dim3(d.Ck, d.SB, pq), kFlashThreads, fl_smem, st>>>(d, Q, Kp, Vp, off_k, ri.goff, ri.pairs, w.o_part, w.l_part);
       MUSE_LAUNCH_OK();
     }
   }
+  prof_mark("k_merge", st);
   k_merge<T, D><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.o_far, w.lse_far, w.o_loc, w.lse_loc, w.o_part, w.l_part, sel, O, LSE);
   MUSE_LAUNCH_OK();
   return MUSE_OK;

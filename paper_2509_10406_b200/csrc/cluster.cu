@@ -66,6 +66,7 @@ k_sort_scan(int32_t* __restrict__ cnt, int nkeys, int nchunks, int32_t* __restri
 }
 
 int launch_scan(int32_t* cnt, int problems, int nkeys, int nchunks, int32_t* off, cudaStream_t st) {
+  prof_mark("k_sort_scan", st);
   k_sort_scan<<<problems, 1024, 0, st>>>(cnt, nkeys, nchunks, off);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
@@ -114,9 +115,11 @@ int bucket_sort(int, const int32_t* assign, int problems, int N, int C, int S, i
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_sort_hist, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_sort_scatter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   }
+  prof_mark("k_sort_hist", st);
   k_sort_hist<<<dim3(nchunks, problems), kSortThreads, smem, st>>>(assign, N, C, S, Bs, kind, nkeys, nchunks, scratch);
   MUSE_LAUNCH_OK();
   if (launch_scan(scratch, problems, nkeys, nchunks, off, st) != MUSE_OK) return MUSE_ERR_CUDA;
+  prof_mark("k_sort_scatter", st);
   k_sort_scatter<<<dim3(nchunks, problems), kSortThreads, smem, st>>>(assign, N, C, S, Bs, kind, nkeys, nchunks, scratch, perm);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
@@ -319,20 +322,24 @@ static int lloyd_t(const Dims& d, const T* X, int problems, int C, int kind, con
   int32_t* perm = ar.take<int32_t>((size_t)problems * d.N);
   int32_t* scratch = ar.take<int32_t>((size_t)problems * sort_ws_elems(d.N, C * d.S));
   if (init_mode != MUSE_INIT_CENTRES) {
+    prof_mark("k_init_centres", st);
     k_init_centres<T><<<dim3(C, problems), 32, 0, st>>>(X, d.N, D, C, init_idx, init_mode, seed, kind, centres);
     MUSE_LAUNCH_OK();
   }
   const int total = problems * C;
+  prof_mark("k_centre_norms", st);
   k_centre_norms<<<cdiv(total * 32, 256), 256, 0, st>>>(centres, total, D, cnorm);
   MUSE_LAUNCH_OK();
   const size_t smem = (size_t)((kAsgRows + kAsgCols) * (D + 4) + kAsgCols) * sizeof(float);
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_assign<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   for (int it = 0; it <= T_iters; ++it) {
+    prof_mark("k_assign", st);
     k_assign<T, D><<<dim3(cdiv(d.N, kAsgRows), problems), kAsgThreads, smem, st>>>(X, d.N, C, centres, cnorm, assign);
     MUSE_LAUNCH_OK();
     if (it == T_iters) break;
     int rc = bucket_sort(0, assign, problems, d.N, C, d.S, d.Bs, kind, off, perm, scratch, st);
     if (rc != MUSE_OK) return rc;
+    prof_mark("k_update", st);
     k_update<T, D><<<dim3(C, problems), 128, 0, st>>>(X, d.N, C, d.S, kind, off, perm, centres, cnorm);
     MUSE_LAUNCH_OK();
   }

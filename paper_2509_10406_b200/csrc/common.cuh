@@ -78,6 +78,9 @@ __device__ __forceinline__ float warp_max(float v) {
   return v;
 }
 
+// per-kernel timing hook (no-op unless muse_profile(1) was called); name = nullptr ends a call
+void prof_mark(const char* name, cudaStream_t st);
+
 // ---- stage launchers (each enqueues on `st`, returns MUSE_OK or MUSE_ERR_CUDA) ---------------
 // clustering side: kind 0 = queries (key = block*C + cluster), kind 1 = keys (key = cluster*S + block)
 size_t sort_ws_elems(int N, int nkeys);   // int32 scratch elements per problem for bucket_sort

@@ -160,14 +160,17 @@ static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const i
   T* Kp = (T*)(base + L.Kp); T* Vp = (T*)(base + L.Vp);
   const int vpr = D * (int)sizeof(T) / 16;
   dim3 gg(cdiv(d.N * vpr, 256), pk);
+  prof_mark("k_gather_rows", st);
   k_gather_rows<T><<<gg, 256, 0, st>>>(K, perm_k, d.N, D, Kp);
   MUSE_LAUNCH_OK();
+  prof_mark("k_gather_rows", st);
   k_gather_rows<T><<<gg, 256, 0, st>>>(V, perm_k, d.N, D, Vp);
   MUSE_LAUNCH_OK();
   if (d.SB == 0) return MUSE_OK;
   const size_t smem = (size_t)(kSumI * (D + 4) + kSumKC * (2 * D + 4) + kSumI * (kSumKC + 1)) * sizeof(float);
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid(d.Ck, cdiv(d.Cq, kSumI), d.B * d.Hq);
+  prof_mark("k_summarize", st);
   k_summarize<T, D><<<grid, kSumThreads, smem, st>>>(d, Kp, Vp, off_k, qbar, (float*)(base + L.mu),
                                                     (float*)(base + L.kappa), (float*)(base + L.nu));
   MUSE_LAUNCH_OK();

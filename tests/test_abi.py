@@ -1,0 +1,74 @@
+"""The C-ABI library builds, loads and exports every symbol include/muse.h declares; host-side
+argument checking works without a GPU (no compute is launched here)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def mb():
+    from paper_2509_10406_b200 import build, binding
+    build.build()
+    binding.lib()
+    return binding
+
+
+def test_header_symbols_are_exported(mb):
+    hdr = open(os.path.join(ROOT, "include", "muse.h")).read()
+    declared = set(re.findall(r"MUSE_API\s+[\w\s\*]+?\b(muse_\w+)\s*\(", hdr))
+    assert declared == set(mb.EXPORTS)
+    lib = ctypes.CDLL(mb.LIB_PATH)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def test_params_struct_layout(mb):
+    assert ctypes.sizeof(mb.MuseParams) == 96
+    assert mb.MuseParams.seed.offset == 64 and mb.MuseParams.head_map.offset == 88
+
+
+def test_workspace_sizes_and_layout(mb):
+    p = mb.make_params(B=1, Hq=16, Hkv=16, N=65536, D=128, Cq=256, Ck=1024, m=32)
+    sizes = mb.muse_workspace_bytes(p)
+    ent = 16 * 7 * 256 * 1024
+    assert sizes[4] >= ent * (2 * 128 + 1) * 4 + 2 * 16 * 65536 * 128 * 2
+    off = mb.muse_summaries_layout(p)
+    assert off[0] == 0 and off[1] >= ent * 4 and off[2] - off[1] >= ent * 128 * 4 and all(o % 256 == 0 for o in off)
+    assert all(s % 256 == 0 for s in sizes)
+
+
+@pytest.mark.parametrize("kw,code", [
+    (dict(D=96), -2), (dict(m=2000), -1), (dict(N=1001), -1), (dict(Cq=0), -1), (dict(k2=1), -2),
+    (dict(dipole=1), -2), (dict(Hq=3, Hkv=2), -1), (dict(m=65, Ck=128), -2), (dict(Ck=8192, N=16384), -2),
+])
+def test_invalid_parameters_are_rejected_on_the_host(mb, kw, code):
+    args = dict(B=1, Hq=2, Hkv=2, N=1024, D=64, Cq=8, Ck=16, m=4)
+    args.update(kw)
+    p = mb.make_params(**args)
+    out = (ctypes.c_size_t * 5)()
+    assert mb.lib().muse_workspace_bytes(ctypes.byref(p), out) == code
+    assert mb.lib().muse_strerror(code)
+
+
+def test_null_and_small_workspace_are_rejected(mb):
+    p = mb.make_params(B=1, Hq=1, Hkv=1, N=1024, D=64, Cq=8, Ck=16, m=4)
+    L = mb.lib()
+    z = ctypes.c_void_p(0)
+    assert L.muse_cluster(ctypes.byref(p), z, z, z, z, z, z, z, z, z, 0, z) == -1
+    fake = ctypes.c_void_p(4096)      # aligned, never dereferenced: the size check comes first
+    assert L.muse_summarize(ctypes.byref(p), fake, fake, fake, fake, fake, fake, fake, fake, 16, z) == -3
+    assert L.muse_attn_fwd(ctypes.byref(p), fake, fake, fake, fake, fake, fake, fake, fake, z, fake, fake, z, fake, 16, z) == -3
+    odd = ctypes.c_void_p(4100)
+    assert L.muse_summarize(ctypes.byref(p), odd, fake, fake, fake, fake, fake, fake, fake, 1 << 30, z) == -1
+
+
+def test_head_map(mb):
+    p = mb.make_params(B=1, Hq=3, Hkv=2, N=1024, D=64, Cq=8, Ck=16, m=4, head_map=[0, 1, 1])
+    assert len(mb.muse_workspace_bytes(p)) == 5
+    p = mb.make_params(B=1, Hq=3, Hkv=2, N=1024, D=64, Cq=8, Ck=16, m=4, head_map=[0, 1, 2])
+    out = (ctypes.c_size_t * 5)()
+    assert mb.lib().muse_workspace_bytes(ctypes.byref(p), out) == -1
