@@ -8,6 +8,10 @@
 namespace muse {
 
 int launch_scan(int32_t* cnt, int problems, int nkeys, int nchunks, int32_t* off, cudaStream_t st);
+int local_fwd_tc(const Dims& d, const void* Q, const void* K, const void* V, float* o_loc, float* lse_loc, int* status,
+                 cudaStream_t st);
+int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
+               const int32_t* pairs, float* o_part, float* l_part, int* status, cudaStream_t st);
 
 // plane of a query = index of the accumulated-summary plane it reads: block - 1 when causal
 // (block 0 sees no far field), 0 when non-causal.
@@ -475,11 +479,12 @@ __global__ void k_merge(Dims dm, const float* __restrict__ o_far, const float* _
 }
 
 // ---------------------------------------------------------------------------------------------
-struct FwdWs { int32_t *off_q, *perm_q, *sort_scratch, *ret_scratch, *sel_tmp; float *o_far, *lse_far, *o_loc, *lse_loc, *o_part, *l_part; };
+struct FwdWs { int32_t *status, *off_q, *perm_q, *sort_scratch, *ret_scratch, *sel_tmp; float *o_far, *lse_far, *o_loc, *lse_loc, *o_part, *l_part; };
 
 static FwdWs fwd_ws(const Dims& d, Arena& ar) {
   FwdWs w;
   const size_t pq = (size_t)d.B * d.Hq;
+  w.status = ar.take<int32_t>(64);          // ws[0]: non-zero if a bounded device-side wait gave up
   w.off_q = ar.take<int32_t>(pq * (d.S * d.Cq + 1));
   w.perm_q = ar.take<int32_t>(pq * d.N);
   w.sort_scratch = ar.take<int32_t>(pq * sort_ws_elems(d.N, d.Cq * d.S));
@@ -508,8 +513,13 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
   const T* Kp = (const T*)(base + L.Kp); const T* Vp = (const T*)(base + L.Vp);
   int32_t* sel = sel_out ? sel_out : w.sel_tmp;
   const size_t fl_smem = 3 * tile_bytes<T, D>() + ptile_bytes();
+  constexpr bool kTensor = sizeof(T) == 2;      // bf16 mode runs the exact-attention parts on tcgen05
+  MUSE_CUDA_OK(cudaMemsetAsync(w.status, 0, 64 * sizeof(int32_t), st));
   // local attention
-  if (d.causal) {
+  if (d.causal && kTensor) {
+    int rc = local_fwd_tc(d, Q, K, V, w.o_loc, w.lse_loc, w.status, st);
+    if (rc != MUSE_OK) return rc;
+  } else if (d.causal) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_local_fwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fl_smem));
     prof_mark("k_local_fwd", st);
     k_local_fwd<T, D><<<dim3(d.S * cdiv(d.Bs, kTile), pq), kFlashThreads, fl_smem, st>>>(d, Q, K, V, w.o_loc, w.lse_loc);
@@ -532,10 +542,15 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
       RetIndex ri;
       rc = build_ret_index(d, sel, w.ret_scratch, &ri, st);
       if (rc != MUSE_OK) return rc;
-      MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fl_smem));
-      prof_mark("k_ret_fwd", st);
-      k_ret_fwd<T, D><<<dim3(d.Ck, d.SB, pq), kFlashThreads, fl_smem, st>>>(d, Q, Kp, Vp, off_k, ri.goff, ri.pairs, w.o_part, w.l_part);
-      MUSE_LAUNCH_OK();
+      if (kTensor) {
+        rc = ret_fwd_tc(d, Q, Kp, Vp, off_k, ri.goff, ri.pairs, w.o_part, w.l_part, w.status, st);
+        if (rc != MUSE_OK) return rc;
+      } else {
+        MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fl_smem));
+        prof_mark("k_ret_fwd", st);
+        k_ret_fwd<T, D><<<dim3(d.Ck, d.SB, pq), kFlashThreads, fl_smem, st>>>(d, Q, Kp, Vp, off_k, ri.goff, ri.pairs, w.o_part, w.l_part);
+        MUSE_LAUNCH_OK();
+      }
     }
   }
   prof_mark("k_merge", st);
