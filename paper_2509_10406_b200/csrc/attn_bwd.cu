@@ -632,14 +632,21 @@ __global__ void k_final_dkv(Dims dm, const int32_t* __restrict__ perm_k, const f
 }
 
 // ---------------------------------------------------------------------------------------------
+int local_bwd_tc(const Dims& d, const void* Q, const void* K, const void* V, const void* dO, const float* LSE,
+                 const float* delta, float* dQacc, float* dK_orig, float* dV_orig, int* status, cudaStream_t st);
+int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, const void* Vp, const float* LSE,
+               const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, float* dq_part,
+               float* dK_perm, float* dV_perm, int* status, cudaStream_t st);
+
 struct BwdWs {
-  int32_t *off_q, *perm_q, *sort_scratch, *ret_scratch;
+  int32_t *status, *off_q, *perm_q, *sort_scratch, *ret_scratch;
   float *delta, *dQacc, *dq_part, *dK_orig, *dV_orig, *dK_perm, *dV_perm, *dkappa, *dnu, *dS;
 };
 
 static BwdWs bwd_ws(const Dims& d, Arena& ar) {
   BwdWs w;
   const size_t pq = (size_t)d.B * d.Hq, ent = pq * d.SB * d.Cq * d.Ck;
+  w.status = ar.take<int32_t>(64);          // ws[0]: non-zero if a bounded device-side wait gave up
   w.off_q = ar.take<int32_t>(pq * (d.S * d.Cq + 1));
   w.perm_q = ar.take<int32_t>(pq * d.N);
   w.sort_scratch = ar.take<int32_t>(pq * sort_ws_elems(d.N, d.Cq * d.S));
@@ -682,7 +689,12 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
   MUSE_CUDA_OK(cudaMemsetAsync(w.dK_perm, 0, nd, st));
   MUSE_CUDA_OK(cudaMemsetAsync(w.dV_perm, 0, nd, st));
   const size_t sm4 = 4 * tile_bytes<T, D>() + ptile_bytes();
-  if (d.causal) {
+  constexpr bool kTensor = sizeof(T) == 2;      // bf16 mode runs the exact-attention parts on tcgen05
+  MUSE_CUDA_OK(cudaMemsetAsync(w.status, 0, 64 * sizeof(int32_t), st));
+  if (d.causal && kTensor) {
+    int rc = local_bwd_tc(d, Q, K, V, dO, LSE, w.delta, w.dQacc, w.dK_orig, w.dV_orig, w.status, st);
+    if (rc != MUSE_OK) return rc;
+  } else if (d.causal) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_local_bwd_dkdv<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm4));
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_local_bwd_dq<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm4));
     dim3 grid(d.S * cdiv(d.Bs, kTile), pq);
@@ -704,11 +716,16 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
       RetIndex ri;
       rc = build_ret_index(d, sel, w.ret_scratch, &ri, st);
       if (rc != MUSE_OK) return rc;
-      MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm4));
-      prof_mark("k_ret_bwd", st);
-      k_ret_bwd<T, D><<<dim3(d.Ck, pq), kFlashThreads, sm4, st>>>(d, Q, dO, Kp, Vp, LSE, w.delta, off_k, ri.goff, ri.pairs,
-                                                                w.dq_part, w.dK_perm, w.dV_perm);
-      MUSE_LAUNCH_OK();
+      if (kTensor) {
+        rc = ret_bwd_tc(d, Q, dO, Kp, Vp, LSE, w.delta, off_k, ri.goff, ri.pairs, w.dq_part, w.dK_perm, w.dV_perm, w.status, st);
+        if (rc != MUSE_OK) return rc;
+      } else {
+        MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm4));
+        prof_mark("k_ret_bwd", st);
+        k_ret_bwd<T, D><<<dim3(d.Ck, pq), kFlashThreads, sm4, st>>>(d, Q, dO, Kp, Vp, LSE, w.delta, off_k, ri.goff, ri.pairs,
+                                                                  w.dq_part, w.dK_perm, w.dV_perm);
+        MUSE_LAUNCH_OK();
+      }
       use_ret = 1;
     }
     const size_t fsm = (size_t)(4 * kTile * (D + 4) + kTile * kLDP) * sizeof(float) + (size_t)kTile * cdiv(d.Ck, 32) * sizeof(uint32_t);

@@ -1,0 +1,455 @@
+// Exact-attention backward on the Blackwell tensor cores (bf16 inputs, fp32 accumulation in
+// tensor memory), for the local block-diagonal component and the retrieved-cluster component.
+// With L the merged log-sum-exp and delta = dO.O (Appendix "Centroid Gradient Flow" fixes what
+// is constant):  P = exp(sigma q.k - L),  G = P (dO.v - delta),
+//                dV = P^T dO,  dK = sigma G^T Q,  dQ = sigma G K.
+// Two tile routines, one thread per accumulator row:
+//   rows-on-M (dQ):      S = Q K^T, dP = dO V^T -> G (bf16, smem) -> dQ += G K      (TMEM)
+//   keys-on-M (dK, dV):  S^T = K Q^T, dP^T = V dO^T -> P^T, G^T -> dV += P^T dO, dK += G^T Q
+// Operand tiles are 128-byte-swizzled in shared memory; a [rows][D] tile serves both as a
+// K-major operand (contraction over D) and as an MN-major operand (contraction over rows).
+#include "common.cuh"
+#include "tc05.cuh"
+
+namespace muse {
+
+typedef __nv_bfloat16 bf16;
+constexpr int kBM = 128, kBN = 64;
+constexpr float kLog2e = 1.4426950408889634f;
+
+template <int D, int ROWS, class RowPtr>
+__device__ __forceinline__ void fill_tile(unsigned char* dst, int n, RowPtr row_ptr, int tid) {
+  constexpr int CPR = D / 8;
+  for (int e = tid; e < ROWS * CPR; e += 128) {
+    const int r = e / CPR, ck = e % CPR, kb = ck >> 3, c = ck & 7;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (r < n) v = reinterpret_cast<const uint4*>(row_ptr(r))[ck];
+    *reinterpret_cast<uint4*>(dst + kb * ROWS * 128 + tc::sw128_off(r, c)) = v;
+  }
+}
+
+// K-major view of a [ROWS][D] tile at k-step ks (16 elements of D)
+template <int ROWS> __device__ __forceinline__ uint64_t desc_k(uint32_t base, int ks) {
+  return tc::smem_desc_sw128(base + (ks / 4) * ROWS * 128 + (ks % 4) * 32, 16, 1024);
+}
+// MN-major view of a [ROWS][D] tile at k-step ks (16 rows)
+template <int ROWS> __device__ __forceinline__ uint64_t desc_mn(uint32_t base, int ks) {
+  return tc::smem_desc_sw128(base + ks * 16 * 128, ROWS * 128, 1024);
+}
+
+struct BwdCtx {
+  unsigned char* sm;
+  uint64_t* bar;
+  uint32_t tbase, ph0, ph1;
+  bool ok;
+};
+
+__device__ __forceinline__ void bwd_setup(BwdCtx& c, unsigned char* sm_raw, uint64_t* bar, uint32_t* tbase_s, uint32_t cols, int tid) {
+  c.sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
+  c.bar = bar; c.ph0 = c.ph1 = 0; c.ok = true;
+  if ((tid >> 5) == 0) tc::tmem_alloc(tbase_s, cols);
+  if (tid == 0) { tc::mbar_init(&bar[0], 1); tc::mbar_init(&bar[1], 1); tc::mbar_init_fence(); }
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  c.tbase = *tbase_s;
+}
+__device__ __forceinline__ void bwd_teardown(BwdCtx& c, uint32_t cols, int tid, int* status) {
+  tc::fence_before_sync();
+  __syncthreads();
+  if ((tid >> 5) == 0) tc::tmem_dealloc(c.tbase, cols);
+  if (!c.ok && tid == 0) atomicExch(status, 2);
+}
+
+__device__ __forceinline__ void store_row64(unsigned char* tile, int row, const float (&x)[kBN]) {
+#pragma unroll
+  for (int ch = 0; ch < kBN / 8; ++ch) {
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      __nv_bfloat162 b = __floats2bfloat162_rn(x[ch * 8 + 2 * k], x[ch * 8 + 2 * k + 1]);
+      w[k] = *reinterpret_cast<uint32_t*>(&b);
+    }
+    *reinterpret_cast<uint4*>(tile + tc::sw128_off(row, ch)) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+// ================================================================================================
+// rows-on-M: dQ of 128 rows (Q, dO tiles already in shared memory) against keys [k_lo, k_hi)
+// ================================================================================================
+template <int D> struct RowsSmem {
+  // the G tile reuses the V tile's bytes: V is dead once the S / dP products have completed
+  static constexpr int q = 0, dO = q + kBM * D * 2, k = dO + kBM * D * 2, v = k + kBN * D * 2, g = v,
+                       total = v + (kBN * D * 2 > kBM * kBN * 2 ? kBN * D * 2 : kBM * kBN * 2) + 1024;
+  static constexpr uint32_t cols = 256;       // S 64 | dP 64 | dQ D
+};
+
+template <int D, class Limit>
+__device__ __forceinline__ bool dq_rows_tc(BwdCtx& c, const bf16* __restrict__ Kb, const bf16* __restrict__ Vb, int k_lo,
+                                           int k_hi, Limit limit, float scale2, float L2, float delta, int tid) {
+  typedef RowsSmem<D> SM;
+  const int warp = tid >> 5;
+  const uint32_t t_s = c.tbase + ((uint32_t)(warp * 32) << 16), t_dp = t_s + kBN;
+  const uint32_t qa = tc::smem_u32(c.sm + SM::q), da = tc::smem_u32(c.sm + SM::dO), ka = tc::smem_u32(c.sm + SM::k),
+                 va = tc::smem_u32(c.sm + SM::v), ga = tc::smem_u32(c.sm + SM::g);
+  const int my_limit = limit(tid);
+  bool first = true;
+  for (int c0 = k_lo; c0 < k_hi && c.ok; c0 += kBN) {
+    const int nk = min(kBN, k_hi - c0);
+    fill_tile<D, kBN>(c.sm + SM::k, nk, [&](int r) { return Kb + (size_t)(c0 + r) * D; }, tid);
+    fill_tile<D, kBN>(c.sm + SM::v, nk, [&](int r) { return Vb + (size_t)(c0 + r) * D; }, tid);
+    tc::fence_async_smem();
+    tc::fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {
+      tc::fence_after_sync();
+      const uint32_t idesc = tc::idesc_bf16(kBM, kBN, 0, 0);
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase, desc_k<kBM>(qa, ks), desc_k<kBN>(ka, ks), idesc, ks > 0);
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase + kBN, desc_k<kBM>(da, ks), desc_k<kBN>(va, ks), idesc, ks > 0);
+      tc::mma_commit(&c.bar[0]);
+    }
+    if (!tc::mbar_wait(&c.bar[0], c.ph0)) { c.ok = false; break; }
+    c.ph0 ^= 1;
+    tc::fence_after_sync();
+    const int vis = min(nk, my_limit - c0 + 1);
+    float g[kBN];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      float s[32], dp[32];
+      tc::tmem_ld32(t_s + 32 * h, s);
+      tc::tmem_ld32(t_dp + 32 * h, dp);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const float p = (32 * h + i) < vis ? exp2f(s[i] * scale2 - L2) : 0.f;
+        g[32 * h + i] = p * (dp[i] - delta);
+      }
+    }
+    store_row64(c.sm + SM::g, tid, g);
+    tc::fence_async_smem();
+    tc::fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {
+      tc::fence_after_sync();
+      const uint32_t idesc = tc::idesc_bf16(kBM, D, 0, 1);
+#pragma unroll
+      for (int ks = 0; ks < kBN / 16; ++ks)
+        tc::mma_bf16_ss(c.tbase + 2 * kBN, tc::smem_desc_sw128(ga + ks * 32, 16, 1024), desc_mn<kBN>(ka, ks), idesc, !(first && ks == 0));
+      tc::mma_commit(&c.bar[1]);
+    }
+    first = false;
+    if (!tc::mbar_wait(&c.bar[1], c.ph1)) { c.ok = false; break; }
+    c.ph1 ^= 1;
+    tc::fence_after_sync();
+  }
+  return !first;          // false: no key tile was processed, the accumulator holds nothing
+}
+
+// Reads this thread's accumulator row (D columns starting at column `col`), scales it by `f`
+// and, if `write`, stores it.  The TMEM load is warp-collective, so EVERY thread of the CTA
+// must call this; only the global store is predicated.
+template <int D>
+__device__ __forceinline__ void read_acc_row(const BwdCtx& c, uint32_t col, float f, float* __restrict__ dst, bool write, int tid) {
+  const uint32_t t = c.tbase + ((uint32_t)((tid >> 5) * 32) << 16) + col;
+#pragma unroll
+  for (int d0 = 0; d0 < D; d0 += 32) {
+    float v[32];
+    tc::tmem_ld32(t + d0, v);
+    if (write) {
+#pragma unroll
+      for (int i = 0; i < 32; i += 4)
+        *reinterpret_cast<float4*>(dst + d0 + i) = make_float4(v[i] * f, v[i + 1] * f, v[i + 2] * f, v[i + 3] * f);
+    }
+  }
+}
+
+template <int D>
+__global__ void __launch_bounds__(128)
+k_local_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ K, const bf16* __restrict__ V,
+                  const bf16* __restrict__ dO, const float* __restrict__ LSE, const float* __restrict__ delta,
+                  float* __restrict__ dQacc, int* __restrict__ status) {
+  extern __shared__ __align__(1024) unsigned char sm_raw[];
+  __shared__ uint64_t bar[2];
+  __shared__ uint32_t tbase_s;
+  const int tid = threadIdx.x;
+  BwdCtx c;
+  bwd_setup(c, sm_raw, bar, &tbase_s, RowsSmem<D>::cols, tid);
+  const int tpb = cdiv(dm.Bs, kBM);
+  const int lin = blockIdx.x, qt = tpb - 1 - lin / dm.S, blk = lin % dm.S, pq = blockIdx.y;
+  const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
+  const int bstart = blk * dm.Bs, bend = bstart + dm.Bs;
+  const int q0 = bstart + qt * kBM, nq = min(kBM, bend - q0);
+  const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
+  const bf16* Kb = K + (size_t)pk * dm.N * D; const bf16* Vb = V + (size_t)pk * dm.N * D;
+  fill_tile<D, kBM>(c.sm + RowsSmem<D>::q, nq, [&](int r) { return Qb + (size_t)(q0 + r) * D; }, tid);
+  fill_tile<D, kBM>(c.sm + RowsSmem<D>::dO, nq, [&](int r) { return dOb + (size_t)(q0 + r) * D; }, tid);
+  const size_t t = (size_t)pq * dm.N + q0 + tid;
+  const float L2 = tid < nq ? LSE[t] * kLog2e : 0.f, dl = tid < nq ? delta[t] : 0.f;
+  dq_rows_tc<D>(c, Kb, Vb, bstart, q0 + nq, [&](int r) { return q0 + r; }, dm.sigma * kLog2e, L2, dl, tid);
+  if (c.ok) read_acc_row<D>(c, 2 * kBN, dm.sigma, dQacc + t * D, tid < nq, tid);
+  bwd_teardown(c, RowsSmem<D>::cols, tid, status);
+}
+
+template <int D>
+__global__ void __launch_bounds__(128)
+k_ret_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO, const bf16* __restrict__ Kp,
+                const bf16* __restrict__ Vp, const float* __restrict__ LSE, const float* __restrict__ delta,
+                const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
+                float* __restrict__ dq_part, int* __restrict__ status) {
+  extern __shared__ __align__(1024) unsigned char sm_raw[];
+  __shared__ uint64_t bar[2];
+  __shared__ uint32_t tbase_s;
+  __shared__ int32_t pid_s[kBM];
+  const int tid = threadIdx.x;
+  const int j = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z;
+  const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
+  const int nkeys = dm.SB * dm.Ck;
+  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)pl * dm.Ck + j;
+  const int g0 = go[0], g1 = go[1];
+  if (g0 >= g1) return;
+  const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
+  const int k0 = ok[0], k1 = ok[pl + 1];
+  BwdCtx c;
+  bwd_setup(c, sm_raw, bar, &tbase_s, RowsSmem<D>::cols, tid);
+  const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
+  const bf16* Kb = Kp + (size_t)pk * dm.N * D; const bf16* Vb = Vp + (size_t)pk * dm.N * D;
+  const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
+  for (int t0 = g0; t0 < g1 && c.ok; t0 += kBM) {
+    const int nq = min(kBM, g1 - t0);
+    __syncthreads();
+    pid_s[tid] = tid < nq ? pr[t0 + tid] : 0;
+    __syncthreads();
+    fill_tile<D, kBM>(c.sm + RowsSmem<D>::q, nq, [&](int r) { return Qb + (size_t)(pid_s[r] / dm.m) * D; }, tid);
+    fill_tile<D, kBM>(c.sm + RowsSmem<D>::dO, nq, [&](int r) { return dOb + (size_t)(pid_s[r] / dm.m) * D; }, tid);
+    const size_t t = (size_t)pq * dm.N + pid_s[tid] / dm.m;
+    const float L2 = tid < nq ? LSE[t] * kLog2e : 0.f, dl = tid < nq ? delta[t] : 0.f;
+    const bool any = dq_rows_tc<D>(c, Kb, Vb, k0, k1, [&](int) { return k1 - 1; }, dm.sigma * kLog2e, L2, dl, tid);
+    if (c.ok) {
+      float* dst = dq_part + ((size_t)pq * dm.N * dm.m + pid_s[tid]) * D;
+      if (any) read_acc_row<D>(c, 2 * kBN, dm.sigma, dst, tid < nq, tid);
+      else if (tid < nq) for (int i = 0; i < D; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    tc::fence_before_sync();
+  }
+  bwd_teardown(c, RowsSmem<D>::cols, tid, status);
+}
+
+// ================================================================================================
+// keys-on-M: dK, dV of 128 keys (K, V tiles already in shared memory), fed 64 query rows at a time
+// ================================================================================================
+template <int D> struct KeysSmem {
+  static constexpr int k = 0, v = k + kBM * D * 2, q = v + kBM * D * 2, dO = q + kBN * D * 2, pt = dO + kBN * D * 2,
+                       gt = pt + kBM * kBN * 2, total = gt + kBM * kBN * 2 + 1024;
+  static constexpr uint32_t cols = D == 128 ? 512 : 256;   // S^T 64 | dP^T 64 | dV D | dK D
+};
+
+// One tile of 64 query rows (already in shared memory with their L2 / delta in Ls / ds).
+// valid(u_row) = number of leading query columns ... see callers: mask(col) tells whether
+// query column `col` sees this thread's key.
+template <int D, class Mask>
+__device__ __forceinline__ void dkdv_step_tc(BwdCtx& c, const float* __restrict__ Ls, const float* __restrict__ ds,
+                                             Mask mask, float scale2, bool& started, int tid) {
+  typedef KeysSmem<D> SM;
+  const int warp = tid >> 5;
+  const uint32_t t_s = c.tbase + ((uint32_t)(warp * 32) << 16), t_dp = t_s + kBN;
+  const uint32_t ka = tc::smem_u32(c.sm + SM::k), va = tc::smem_u32(c.sm + SM::v), qa = tc::smem_u32(c.sm + SM::q),
+                 da = tc::smem_u32(c.sm + SM::dO), pa = tc::smem_u32(c.sm + SM::pt), ga = tc::smem_u32(c.sm + SM::gt);
+  tc::fence_async_smem();
+  tc::fence_before_sync();
+  __syncthreads();
+  if (tid == 0) {
+    tc::fence_after_sync();
+    const uint32_t idesc = tc::idesc_bf16(kBM, kBN, 0, 0);
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase, desc_k<kBM>(ka, ks), desc_k<kBN>(qa, ks), idesc, ks > 0);
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase + kBN, desc_k<kBM>(va, ks), desc_k<kBN>(da, ks), idesc, ks > 0);
+    tc::mma_commit(&c.bar[0]);
+  }
+  if (!tc::mbar_wait(&c.bar[0], c.ph0)) { c.ok = false; return; }
+  c.ph0 ^= 1;
+  tc::fence_after_sync();
+  float p[kBN], g[kBN];
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    float s[32], dp[32];
+    tc::tmem_ld32(t_s + 32 * h, s);
+    tc::tmem_ld32(t_dp + 32 * h, dp);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const int col = 32 * h + i;
+      const float pv = mask(col) ? exp2f(s[i] * scale2 - Ls[col]) : 0.f;
+      p[col] = pv;
+      g[col] = pv * (dp[i] - ds[col]);
+    }
+  }
+  store_row64(c.sm + SM::pt, tid, p);
+  store_row64(c.sm + SM::gt, tid, g);
+  tc::fence_async_smem();
+  tc::fence_before_sync();
+  __syncthreads();
+  if (tid == 0) {
+    tc::fence_after_sync();
+    const uint32_t idesc = tc::idesc_bf16(kBM, D, 0, 1);
+#pragma unroll
+    for (int ks = 0; ks < kBN / 16; ++ks)
+      tc::mma_bf16_ss(c.tbase + 2 * kBN, tc::smem_desc_sw128(pa + ks * 32, 16, 1024), desc_mn<kBN>(da, ks), idesc, !(!started && ks == 0));
+#pragma unroll
+    for (int ks = 0; ks < kBN / 16; ++ks)
+      tc::mma_bf16_ss(c.tbase + 2 * kBN + D, tc::smem_desc_sw128(ga + ks * 32, 16, 1024), desc_mn<kBN>(qa, ks), idesc, !(!started && ks == 0));
+    tc::mma_commit(&c.bar[1]);
+  }
+  started = true;
+  if (!tc::mbar_wait(&c.bar[1], c.ph1)) { c.ok = false; return; }
+  c.ph1 ^= 1;
+  tc::fence_after_sync();
+}
+
+template <int D>
+__global__ void __launch_bounds__(128)
+k_local_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ K, const bf16* __restrict__ V,
+                    const bf16* __restrict__ dO, const float* __restrict__ LSE, const float* __restrict__ delta,
+                    float* __restrict__ dK_orig, float* __restrict__ dV_orig, int* __restrict__ status) {
+  typedef KeysSmem<D> SM;
+  extern __shared__ __align__(1024) unsigned char sm_raw[];
+  __shared__ uint64_t bar[2];
+  __shared__ uint32_t tbase_s;
+  __shared__ float Ls[kBN], ds[kBN];
+  const int tid = threadIdx.x;
+  BwdCtx c;
+  bwd_setup(c, sm_raw, bar, &tbase_s, SM::cols, tid);
+  const int tpb = cdiv(dm.Bs, kBM);
+  const int lin = blockIdx.x, kt = lin / dm.S, blk = lin % dm.S, pq = blockIdx.y;   // early key tiles (most work) first
+  const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
+  const int bstart = blk * dm.Bs, bend = bstart + dm.Bs;
+  const int k0 = bstart + kt * kBM, nk = min(kBM, bend - k0);
+  const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
+  const bf16* Kb = K + (size_t)pk * dm.N * D; const bf16* Vb = V + (size_t)pk * dm.N * D;
+  fill_tile<D, kBM>(c.sm + SM::k, nk, [&](int r) { return Kb + (size_t)(k0 + r) * D; }, tid);
+  fill_tile<D, kBM>(c.sm + SM::v, nk, [&](int r) { return Vb + (size_t)(k0 + r) * D; }, tid);
+  bool started = false;
+  const int u = k0 + tid;
+  for (int q0 = k0; q0 < bend && c.ok; q0 += kBN) {
+    const int nq = min(kBN, bend - q0);
+    fill_tile<D, kBN>(c.sm + SM::q, nq, [&](int r) { return Qb + (size_t)(q0 + r) * D; }, tid);
+    fill_tile<D, kBN>(c.sm + SM::dO, nq, [&](int r) { return dOb + (size_t)(q0 + r) * D; }, tid);
+    if (tid < kBN) {
+      Ls[tid] = tid < nq ? LSE[(size_t)pq * dm.N + q0 + tid] * kLog2e : 0.f;
+      ds[tid] = tid < nq ? delta[(size_t)pq * dm.N + q0 + tid] : 0.f;
+    }
+    dkdv_step_tc<D>(c, Ls, ds, [&](int col) { return col < nq && tid < nk && u <= q0 + col; }, dm.sigma * kLog2e, started, tid);
+  }
+  if (c.ok) {
+    const size_t row = ((size_t)pq * dm.N + k0 + tid) * D;
+    read_acc_row<D>(c, 2 * kBN, 1.f, dV_orig + row, tid < nk, tid);
+    read_acc_row<D>(c, 2 * kBN + D, dm.sigma, dK_orig + row, tid < nk, tid);
+  }
+  bwd_teardown(c, SM::cols, tid, status);
+}
+
+// One CTA per (key cluster j, head): 128-key tiles of the cluster's visible run; every plane that
+// sees a tile feeds its retrieving pairs 64 at a time.
+template <int D>
+__global__ void __launch_bounds__(128)
+k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO, const bf16* __restrict__ Kp,
+                  const bf16* __restrict__ Vp, const float* __restrict__ LSE, const float* __restrict__ delta,
+                  const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
+                  float* __restrict__ dK_perm, float* __restrict__ dV_perm, int* __restrict__ status) {
+  typedef KeysSmem<D> SM;
+  extern __shared__ __align__(1024) unsigned char sm_raw[];
+  __shared__ uint64_t bar[2];
+  __shared__ uint32_t tbase_s;
+  __shared__ float Ls[kBN], ds[kBN];
+  __shared__ int32_t tok_s[kBN];
+  const int tid = threadIdx.x;
+  const int j = blockIdx.x, pq = blockIdx.y;
+  const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
+  const int nkeys = dm.SB * dm.Ck;
+  const int32_t* go = goff + (size_t)pq * (nkeys + 1);
+  const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
+  const int kbeg = ok[0], kvis = ok[dm.SB];
+  int total_pairs = 0;
+  for (int pl = 0; pl < dm.SB; ++pl) total_pairs += go[(size_t)pl * dm.Ck + j + 1] - go[(size_t)pl * dm.Ck + j];
+  if (kbeg >= kvis || total_pairs == 0) return;
+  BwdCtx c;
+  bwd_setup(c, sm_raw, bar, &tbase_s, SM::cols, tid);
+  const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
+  const bf16* Kb = Kp + (size_t)pk * dm.N * D; const bf16* Vb = Vp + (size_t)pk * dm.N * D;
+  const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
+  for (int c0 = kbeg; c0 < kvis && c.ok; c0 += kBM) {
+    const int nkc = min(kBM, kvis - c0);
+    __syncthreads();
+    fill_tile<D, kBM>(c.sm + SM::k, nkc, [&](int r) { return Kb + (size_t)(c0 + r) * D; }, tid);
+    fill_tile<D, kBM>(c.sm + SM::v, nkc, [&](int r) { return Vb + (size_t)(c0 + r) * D; }, tid);
+    bool started = false;
+    for (int pl = 0; pl < dm.SB && c.ok; ++pl) {
+      const int vis_end = ok[pl + 1];
+      if (c0 >= vis_end) continue;
+      const bool mine = c0 + tid < vis_end;                // this thread's key is visible to the plane
+      const int g0 = go[(size_t)pl * dm.Ck + j], g1 = go[(size_t)pl * dm.Ck + j + 1];
+      for (int t0 = g0; t0 < g1 && c.ok; t0 += kBN) {
+        const int nq = min(kBN, g1 - t0);
+        __syncthreads();
+        if (tid < kBN) {
+          const int tok = tid < nq ? pr[t0 + tid] / dm.m : 0;
+          tok_s[tid] = tok;
+          Ls[tid] = tid < nq ? LSE[(size_t)pq * dm.N + tok] * kLog2e : 0.f;
+          ds[tid] = tid < nq ? delta[(size_t)pq * dm.N + tok] : 0.f;
+        }
+        __syncthreads();
+        fill_tile<D, kBN>(c.sm + SM::q, nq, [&](int r) { return Qb + (size_t)tok_s[r] * D; }, tid);
+        fill_tile<D, kBN>(c.sm + SM::dO, nq, [&](int r) { return dOb + (size_t)tok_s[r] * D; }, tid);
+        dkdv_step_tc<D>(c, Ls, ds, [&](int col) { return col < nq && mine; }, dm.sigma * kLog2e, started, tid);
+      }
+    }
+    if (c.ok && started) {
+      const size_t row = ((size_t)pq * dm.N + c0 + tid) * D;
+      read_acc_row<D>(c, 2 * kBN, 1.f, dV_perm + row, tid < nkc, tid);
+      read_acc_row<D>(c, 2 * kBN + D, dm.sigma, dK_perm + row, tid < nkc, tid);
+    }
+    tc::fence_before_sync();
+  }
+  bwd_teardown(c, SM::cols, tid, status);
+}
+
+// ---- launchers ------------------------------------------------------------------------------------
+#define MUSE_TC_LAUNCH(KERNEL, SMEM, GRID, ...)                                                                   \
+  do {                                                                                                            \
+    if (d.D == 128) {                                                                                             \
+      MUSE_CUDA_OK(cudaFuncSetAttribute(KERNEL<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM<128>::total)); \
+      KERNEL<128><<<GRID, 128, SMEM<128>::total, st>>>(__VA_ARGS__);                                              \
+    } else {                                                                                                      \
+      MUSE_CUDA_OK(cudaFuncSetAttribute(KERNEL<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM<64>::total));   \
+      KERNEL<64><<<GRID, 128, SMEM<64>::total, st>>>(__VA_ARGS__);                                                \
+    }                                                                                                             \
+    MUSE_LAUNCH_OK();                                                                                             \
+  } while (0)
+
+int local_bwd_tc(const Dims& d, const void* Q, const void* K, const void* V, const void* dO, const float* LSE,
+                 const float* delta, float* dQacc, float* dK_orig, float* dV_orig, int* status, cudaStream_t st) {
+  const int pq = d.B * d.Hq;
+  dim3 grid(d.S * cdiv(d.Bs, kBM), pq);
+  prof_mark("k_local_bwd_dkdv_tc", st);
+  MUSE_TC_LAUNCH(k_local_bwd_dkdv_tc, KeysSmem, grid, d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, (const bf16*)dO, LSE,
+                 delta, dK_orig, dV_orig, status);
+  prof_mark("k_local_bwd_dq_tc", st);
+  MUSE_TC_LAUNCH(k_local_bwd_dq_tc, RowsSmem, grid, d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, (const bf16*)dO, LSE,
+                 delta, dQacc, status);
+  return MUSE_OK;
+}
+
+int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, const void* Vp, const float* LSE,
+               const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, float* dq_part,
+               float* dK_perm, float* dV_perm, int* status, cudaStream_t st) {
+  const int pq = d.B * d.Hq;
+  prof_mark("k_ret_bwd_dkdv_tc", st);
+  MUSE_TC_LAUNCH(k_ret_bwd_dkdv_tc, KeysSmem, dim3(d.Ck, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
+                 (const bf16*)Vp, LSE, delta, off_k, goff, pairs, dK_perm, dV_perm, status);
+  prof_mark("k_ret_bwd_dq_tc", st);
+  MUSE_TC_LAUNCH(k_ret_bwd_dq_tc, RowsSmem, dim3(d.Ck, d.SB, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
+                 (const bf16*)Vp, LSE, delta, off_k, goff, pairs, dq_part, status);
+  return MUSE_OK;
+}
+
+}  // namespace muse
