@@ -81,15 +81,22 @@ typedef struct muse_params {
 /* Sizes in bytes of the scratch each stage needs and of the opaque summaries buffer.
  * out[0] cluster, out[1] summarize, out[2] attn_fwd, out[3] attn_bwd, out[4] summaries.
  * Appendix "Clustering Cost" / Section "Summary Computation": the summaries buffer holds the
- * S-1 accumulated (mu, kappa, nu) planes, [B,Hq,S-1,Cq,Ck] x (1 + 2D) fp32, followed by the
- * bucketed copies of K and V. */
+ * S-1 accumulated (mu, beta, kappa, nu) planes over [B,Hq,S-1,Cq,Ck], followed by the bucketed
+ * copies of K and V (see muse_summaries_layout). */
 MUSE_API int muse_workspace_bytes(const muse_params_t* p, size_t out[5]);
 
-/* Byte offsets inside the summaries buffer: off[0] mu [B,Hq,SB,Cq,Ck] f32, off[1] kappa
- * [B,Hq,SB,Cq,Ck,D] f32, off[2] nu (same), off[3] K bucketed [B,Hkv,N,D] dtype, off[4] V
- * bucketed; SB = S-1 (causal) or 1.  Plane s of mu/kappa/nu is the accumulated summary seen
- * by queries of block s+1 (Section "Causal accumulation": exclusive, block 0 sees nothing). */
-MUSE_API int muse_summaries_layout(const muse_params_t* p, size_t off[5]);
+/* Byte offsets inside the summaries buffer, per entry e = (b, h, plane, i, j) of
+ * [B,Hq,SB,Cq,Ck], SB = S-1 (causal) or 1; plane s is the accumulated summary seen by queries
+ * of block s+1 (Section "Causal accumulation": exclusive, block 0 sees nothing):
+ *   off[0] mu    f32 [e]    accumulated log-mass, -inf for a cluster with no visible key
+ *   off[1] beta  f32 [e]    mu - sigma qbar_i . kappa, so that the Eq. 6 score of a query q is
+ *                           sigma q . kappa + beta
+ *   off[2] kappa     [e][D] fp32 mode: fp32.  bf16 mode: the bf16 rounding of kappa ...
+ *   off[3] kappa_lo  [e][D] ... and the bf16 rounding of the remainder (kappa = hi + lo);
+ *                           fp32 mode: unused (same offset as off[4])
+ *   off[4] nu        [e][D] fp32 (fp32 mode) or bf16 (bf16 mode)
+ *   off[5], off[6]          K and V bucketed by (cluster, block), [B,Hkv,N,D] dtype */
+MUSE_API int muse_summaries_layout(const muse_params_t* p, size_t off[7]);
 
 /* Lloyd k-means of the queries (per query head, Cq clusters) and keys (per kv head, Ck
  * clusters): T x (assign to argmin_c |c|^2 - 2 x.c, lowest index on ties; move each centre to

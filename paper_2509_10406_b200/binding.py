@@ -137,7 +137,8 @@ def muse_profile_report() -> dict:
 
 
 def muse_summaries_layout(p: MuseParams):
-    out = (ctypes.c_size_t * 5)()
+    """Byte offsets (mu, beta, kappa, kappa_lo, nu, K bucketed, V bucketed)."""
+    out = (ctypes.c_size_t * 7)()
     _check(lib().muse_summaries_layout(ctypes.byref(p), out), "muse_summaries_layout")
     return tuple(int(x) for x in out)
 
@@ -193,15 +194,20 @@ class MuseBuffers:
             self.dQ = e(B, Hq, N, D, dtype=dt); self.dK = e(B, Hkv, N, D, dtype=dt); self.dV = e(B, Hkv, N, D, dtype=dt)
 
     def summary_planes(self):
-        """Views (mu, kappa, nu) of the accumulated summaries: [B,Hq,SB,Cq,Ck(,D)] fp32."""
+        """(mu, beta, kappa, nu) of the accumulated summaries as fp32 tensors
+        [B,Hq,SB,Cq,Ck(,D)]; in bf16 mode kappa is rebuilt as hi + lo."""
         p = self.p
         off = muse_summaries_layout(p)
         ent = p.B * p.Hq * p.SB * p.Cq * p.Ck
-        f = lambda o, n: self.summaries[o:o + 4 * n].view(torch.float32)
-        mu = f(off[0], ent).view(p.B, p.Hq, p.SB, p.Cq, p.Ck)
-        ka = f(off[1], ent * p.D).view(p.B, p.Hq, p.SB, p.Cq, p.Ck, p.D)
-        nu = f(off[2], ent * p.D).view(p.B, p.Hq, p.SB, p.Cq, p.Ck, p.D)
-        return mu, ka, nu
+        shp = (p.B, p.Hq, p.SB, p.Cq, p.Ck)
+        f32 = lambda o, n: self.summaries[o:o + 4 * n].view(torch.float32)
+        b16 = lambda o, n: self.summaries[o:o + 2 * n].view(torch.bfloat16).float()
+        mu, beta = f32(off[0], ent).view(shp), f32(off[1], ent).view(shp)
+        if p.dtype == MUSE_F32:
+            ka, nu = f32(off[2], ent * p.D), f32(off[4], ent * p.D)
+        else:
+            ka, nu = b16(off[2], ent * p.D) + b16(off[3], ent * p.D), b16(off[4], ent * p.D)
+        return mu, beta, ka.view(*shp, p.D), nu.view(*shp, p.D)
 
 
 def muse_layer_forward(p, buf: MuseBuffers, Q, K, V, init_q=None, init_k=None, sel_in=None):

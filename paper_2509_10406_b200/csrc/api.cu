@@ -70,13 +70,13 @@ int muse_workspace_bytes(const muse_params_t* p, size_t out[5]) {
   return MUSE_OK;
 }
 
-int muse_summaries_layout(const muse_params_t* p, size_t off[5]) {
+int muse_summaries_layout(const muse_params_t* p, size_t off[7]) {
   Dims d;
   int rc = resolve(p, &d);
   if (rc != MUSE_OK) return rc;
   if (off == nullptr) return MUSE_ERR_INVALID_ARG;
   SummLayout L = summ_layout(d, p->dtype);
-  off[0] = L.mu; off[1] = L.kappa; off[2] = L.nu; off[3] = L.Kp; off[4] = L.Vp;
+  off[0] = L.mu; off[1] = L.beta; off[2] = L.khi; off[3] = L.klo; off[4] = L.nu; off[5] = L.Kp; off[6] = L.Vp;
   return MUSE_OK;
 }
 

@@ -300,8 +300,7 @@ template <class T, int D>
 __global__ void __launch_bounds__(kFlashThreads)
 k_far_bwd(Dims dm, const T* __restrict__ Q, const T* __restrict__ dO, const float* __restrict__ qbar,
           const float* __restrict__ LSE, const float* __restrict__ delta, const int32_t* __restrict__ off_q,
-          const int32_t* __restrict__ perm_q, const int32_t* __restrict__ sel, const float* __restrict__ mu,
-          const float* __restrict__ kappa, const float* __restrict__ nu, float* __restrict__ dQacc,
+          const int32_t* __restrict__ perm_q, const int32_t* __restrict__ sel, SummPtrs sp, float* __restrict__ dQacc,
           float* __restrict__ dkappa, float* __restrict__ dnu, float* __restrict__ dS) {
   constexpr int LD = D + 4;
   extern __shared__ __align__(16) unsigned char smraw[];
@@ -358,11 +357,11 @@ k_far_bwd(Dims dm, const T* __restrict__ Q, const T* __restrict__ dO, const floa
     for (int e = tid; e < kTile * (D / 4); e += kFlashThreads) {
       const int r = e / (D / 4), q = e % (D / 4);
       float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-      if (j0 + r < Ck) { a = ld4(kappa + (ent0 + j0 + r) * D + q * 4); b = ld4(nu + (ent0 + j0 + r) * D + q * 4); }
+      if (j0 + r < Ck) { a = ld_kappa4<T>(sp, (ent0 + j0 + r) * D + q * 4); b = ld_nu4<T>(sp, (ent0 + j0 + r) * D + q * 4); }
       st4(kap + r * LD + q * 4, a);
       st4(nus + r * LD + q * 4, b);
     }
-    if (tid < kTile) mus[tid] = j0 + tid < Ck ? mu[ent0 + j0 + tid] : -INFINITY;
+    if (tid < kTile) mus[tid] = j0 + tid < Ck ? sp.mu[ent0 + j0 + tid] : -INFINITY;
     float dka[4][D / 64][4], dnv[4][D / 64][4];
     float dmu_acc = 0.f;                               // threads 0..63: column tid
     zero_acc<D>(dka); zero_acc<D>(dnv);
@@ -677,9 +676,8 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
   SummLayout L = summ_layout(d, dtype);
   const char* base = (const char*)summaries;
   const T* Kp = (const T*)(base + L.Kp); const T* Vp = (const T*)(base + L.Vp);
-  const float* mu = (const float*)(base + L.mu);
-  const float* kappa = (const float*)(base + L.kappa);
-  const float* nu = (const float*)(base + L.nu);
+  const SummPtrs sp = summ_ptrs(L, base);
+  const float* mu = sp.mu;
   const size_t nd = (size_t)pq * d.N * d.D * sizeof(float);
   const long long rows = (long long)pq * d.N;
   prof_mark("k_delta", st);
@@ -731,8 +729,8 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
     const size_t fsm = (size_t)(4 * kTile * (D + 4) + kTile * kLDP) * sizeof(float) + (size_t)kTile * cdiv(d.Ck, 32) * sizeof(uint32_t);
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fsm));
     prof_mark("k_far_bwd", st);
-    k_far_bwd<T, D><<<dim3(d.Cq, d.SB, pq), kFlashThreads, fsm, st>>>(d, Q, dO, qbar, LSE, w.delta, w.off_q, w.perm_q, sel, mu,
-                                                                    kappa, nu, w.dQacc, w.dkappa, w.dnu, w.dS);
+    k_far_bwd<T, D><<<dim3(d.Cq, d.SB, pq), kFlashThreads, fsm, st>>>(d, Q, dO, qbar, LSE, w.delta, w.off_q, w.perm_q, sel, sp,
+                                                                    w.dQacc, w.dkappa, w.dnu, w.dS);
     MUSE_LAUNCH_OK();
     const size_t ssm = (size_t)(5 * kTile * (D + 4) + kTile * kLDP) * sizeof(float);
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));

@@ -4,12 +4,16 @@
 // and the log-sum-exp merge ("Output merging").
 #include "common.cuh"
 #include "flash_core.cuh"
+#include <cstdlib>
 
 namespace muse {
 
 int launch_scan(int32_t* cnt, int problems, int nkeys, int nchunks, int32_t* off, cudaStream_t st);
 int local_fwd_tc(const Dims& d, const void* Q, const void* K, const void* V, float* o_loc, float* lse_loc, int* status,
                  cudaStream_t st);
+bool far_fwd_tc_supported(const Dims& d, int dtype);
+int far_fwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const int32_t* off_q, const int32_t* perm_q,
+               const int32_t* sel_in, int32_t* sel_out, float* o_far, float* lse_far, int* status, cudaStream_t st);
 int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
                const int32_t* pairs, float* o_part, float* l_part, int* status, cudaStream_t st);
 
@@ -85,8 +89,7 @@ __host__ __device__ inline int far_rows(int Ck) { return Ck <= 1024 ? 32 : Ck <=
 template <class T, int D>
 __global__ void __launch_bounds__(kFarThreads)
 k_far_fwd(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, const int32_t* __restrict__ off_q,
-          const int32_t* __restrict__ perm_q, const float* __restrict__ mu, const float* __restrict__ kappa,
-          const float* __restrict__ nu, const int32_t* __restrict__ sel_in, int32_t* __restrict__ sel_out,
+          const int32_t* __restrict__ perm_q, SummPtrs sp, const int32_t* __restrict__ sel_in, int32_t* __restrict__ sel_out,
           float* __restrict__ o_far, float* __restrict__ lse_far) {
   constexpr int LD = D + 4;
   const int RT = far_rows(dm.Ck), Ck = dm.Ck, LDS_ = Ck + 4;
@@ -104,9 +107,7 @@ k_far_fwd(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, cons
   const int p0 = oq[0], p1 = oq[1];
   if (p0 >= p1) return;
   const size_t ent0 = (((size_t)pq * dm.SB + pl) * dm.Cq + i) * Ck;
-  const float* mup = mu + ent0;
-  const float* kap = kappa + ent0 * D;
-  const float* nup = nu + ent0 * D;
+  const float* mup = sp.mu + ent0;
   const T* Qp = Q + (size_t)pq * dm.N * D;
   const float* qb = qbar + ((size_t)pq * dm.Cq + i) * D;
   const int32_t* pm = perm_q + (size_t)pq * dm.N;
@@ -153,7 +154,7 @@ k_far_fwd(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, cons
       for (int e = tid; e < kFarJC * (D / 4); e += kFarThreads) {
         int r = e / (D / 4), q = e % (D / 4);
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (j0 + r < Ck) v = ld4(kap + (size_t)(j0 + r) * D + q * 4);
+        if (j0 + r < Ck) v = ld_kappa4<T>(sp, (ent0 + j0 + r) * D + q * 4);
         st4(ch + r * LD + q * 4, v);
       }
       __syncthreads();
@@ -239,7 +240,7 @@ k_far_fwd(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, cons
       for (int e = tid; e < kFarJC * (D / 4); e += kFarThreads) {
         int r = e / (D / 4), q = e % (D / 4);
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (j0 + r < Ck) v = ld4(nup + (size_t)(j0 + r) * D + q * 4);
+        if (j0 + r < Ck) v = ld_nu4<T>(sp, (ent0 + j0 + r) * D + q * 4);
         st4(ch + r * LD + q * 4, v);
       }
       __syncthreads();
@@ -531,13 +532,17 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
   if (d.SB > 0) {
     int rc = bucket_sort(0, assign_q, pq, d.N, d.Cq, d.S, d.Bs, 0, w.off_q, w.perm_q, w.sort_scratch, st);
     if (rc != MUSE_OK) return rc;
-    const size_t fs = far_smem(d.Ck, D);
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_fwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fs));
-    prof_mark("k_far_fwd", st);
-    k_far_fwd<T, D><<<dim3(d.Cq, d.SB, pq), kFarThreads, fs, st>>>(
-        d, Q, qbar, w.off_q, w.perm_q, (const float*)(base + L.mu), (const float*)(base + L.kappa),
-        (const float*)(base + L.nu), sel_in, sel, w.o_far, w.lse_far);
-    MUSE_LAUNCH_OK();
+    if (far_fwd_tc_supported(d, dtype) && getenv("MUSE_FAR_SIMT") == nullptr) {
+      rc = far_fwd_tc(d, summ_ptrs(L, base), Q, w.off_q, w.perm_q, sel_in, sel, w.o_far, w.lse_far, w.status, st);
+      if (rc != MUSE_OK) return rc;
+    } else {
+      const size_t fs = far_smem(d.Ck, D);
+      MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_fwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fs));
+      prof_mark("k_far_fwd", st);
+      k_far_fwd<T, D><<<dim3(d.Cq, d.SB, pq), kFarThreads, fs, st>>>(
+          d, Q, qbar, w.off_q, w.perm_q, summ_ptrs(L, base), sel_in, sel, w.o_far, w.lse_far);
+      MUSE_LAUNCH_OK();
+    }
     if (d.m > 0) {
       RetIndex ri;
       rc = build_ret_index(d, sel, w.ret_scratch, &ri, st);

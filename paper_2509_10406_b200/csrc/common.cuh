@@ -97,8 +97,44 @@ int summarize(const Dims& d, int dtype, const void* K, const void* V, const int3
               cudaStream_t st);
 size_t summarize_ws_bytes(const Dims& d);
 
-struct SummLayout { size_t mu, kappa, nu, Kp, Vp, total; };
+// Byte offsets inside the caller's summaries buffer.  Per entry (b, h, plane, i, j):
+//   mu   fp32  accumulated log-mass            beta fp32  mu - sigma qbar_i . kappa  (so that the
+//   Eq. 6 score is sigma q . kappa + beta with the full query)
+//   fp32 mode: kappa, nu fp32 [D]   (klo unused)
+//   bf16 mode: kappa = khi + klo, two bf16 planes [D] (tensor-core operands that keep ~16 bits
+//              of mantissa, so discrete top-m decisions match fp64); nu one bf16 plane [D]
+struct SummLayout { size_t mu, beta, khi, klo, nu, Kp, Vp, total; };
 SummLayout summ_layout(const Dims& d, int dtype);
+
+struct SummPtrs { float* mu; float* beta; void* khi; void* klo; void* nu; };
+inline SummPtrs summ_ptrs(const SummLayout& L, const void* base_) {
+  char* b = (char*)base_;
+  return SummPtrs{(float*)(b + L.mu), (float*)(b + L.beta), b + L.khi, b + L.klo, b + L.nu};
+}
+// ST = storage element type of kappa / nu (float or bf16); idx = element index (entry * D + d), d % 4 == 0
+template <class ST> __device__ __forceinline__ float4 ld_kappa4(const SummPtrs& s, size_t idx);
+template <> __device__ __forceinline__ float4 ld_kappa4<float>(const SummPtrs& s, size_t idx) { return ld4((const float*)s.khi + idx); }
+template <> __device__ __forceinline__ float4 ld_kappa4<__nv_bfloat16>(const SummPtrs& s, size_t idx) {
+  float4 a = ld4((const __nv_bfloat16*)s.khi + idx), b = ld4((const __nv_bfloat16*)s.klo + idx);
+  return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+}
+// value that the stored kappa represents: x itself (fp32) or hi + lo (two bf16)
+template <class ST> __device__ __forceinline__ float kappa_repr(float x);
+template <> __device__ __forceinline__ float kappa_repr<float>(float x) { return x; }
+template <> __device__ __forceinline__ float kappa_repr<__nv_bfloat16>(float x) {
+  const float h = __bfloat162float(__float2bfloat16_rn(x));
+  return h + __bfloat162float(__float2bfloat16_rn(x - h));
+}
+template <class ST> __device__ __forceinline__ float4 ld_nu4(const SummPtrs& s, size_t idx) { return ld4((const ST*)s.nu + idx); }
+template <class ST> __device__ __forceinline__ void st_kappa4(const SummPtrs& s, size_t idx, float4 v);
+template <> __device__ __forceinline__ void st_kappa4<float>(const SummPtrs& s, size_t idx, float4 v) { st4((float*)s.khi + idx, v); }
+template <> __device__ __forceinline__ void st_kappa4<__nv_bfloat16>(const SummPtrs& s, size_t idx, float4 v) {
+  const float hx = __bfloat162float(__float2bfloat16_rn(v.x)), hy = __bfloat162float(__float2bfloat16_rn(v.y)),
+              hz = __bfloat162float(__float2bfloat16_rn(v.z)), hw = __bfloat162float(__float2bfloat16_rn(v.w));
+  st4((__nv_bfloat16*)s.khi + idx, make_float4(hx, hy, hz, hw));
+  st4((__nv_bfloat16*)s.klo + idx, make_float4(v.x - hx, v.y - hy, v.z - hz, v.w - hw));
+}
+template <class ST> __device__ __forceinline__ void st_nu4(const SummPtrs& s, size_t idx, float4 v) { st4((ST*)s.nu + idx, v); }
 
 int attn_fwd(const Dims& d, int dtype, const void* Q, const void* K, const void* V,
              const int32_t* assign_q, const float* qbar, const int32_t* off_k, const int32_t* perm_k,

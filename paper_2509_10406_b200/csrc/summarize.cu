@@ -11,9 +11,11 @@ SummLayout summ_layout(const Dims& d, int dtype) {
   auto up = [](size_t x) { return (x + 255) & ~size_t(255); };
   SummLayout L;
   L.mu = 0;
-  L.kappa = up(L.mu + ent * sizeof(float));
-  L.nu = up(L.kappa + ent * d.D * sizeof(float));
-  L.Kp = up(L.nu + ent * d.D * sizeof(float));
+  L.beta = up(L.mu + ent * sizeof(float));
+  L.khi = up(L.beta + ent * sizeof(float));
+  L.klo = up(L.khi + ent * d.D * es);
+  L.nu = dtype == MUSE_F32 ? L.klo : up(L.klo + ent * d.D * es);
+  L.Kp = up(L.nu + ent * d.D * es);
   L.Vp = up(L.Kp + (size_t)d.B * d.Hkv * d.N * d.D * es);
   L.total = up(L.Vp + (size_t)d.B * d.Hkv * d.N * d.D * es);
   return L;
@@ -42,8 +44,7 @@ constexpr int kSumI = 64, kSumKC = 16, kSumThreads = 256;
 template <class T, int D>
 __global__ void __launch_bounds__(kSumThreads)
 k_summarize(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const int32_t* __restrict__ off_k,
-            const float* __restrict__ qbar, float* __restrict__ mu, float* __restrict__ kappa,
-            float* __restrict__ nu) {
+            const float* __restrict__ qbar, SummPtrs sp) {
   constexpr int LDQ = D + 4, LDKV = 2 * D + 4, LDL = kSumKC + 1, NV = 2 * D / 32;
   extern __shared__ float smf[];
   float* qb = smf;                         // [64][LDQ]  sigma * qbar tile
@@ -132,17 +133,29 @@ k_summarize(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const i
 #pragma unroll
     for (int a = 0; a < 2; ++a) {
       const int i = i0 + ip * 2 + a;
-      if (i >= dm.Cq) continue;
+      const bool live = i < dm.Cq;          // no early exit: the shuffles below need the whole warp
       const size_t ent = (((size_t)pq * dm.SB + b) * dm.Cq + i) * dm.Ck + j;
       const bool some = s[a] > 0.f;
       const float inv = some ? 1.f / s[a] : 0.f;
-      if (sl == 0) mu[ent] = some ? M[a] + logf(s[a]) : -INFINITY;
+      // beta = mu - sigma qbar_i . kappa: partial dot over this thread's kappa dims, summed over the 8 slices
+      float qk = 0.f;
 #pragma unroll
       for (int k = 0; k < NV; ++k) {
         const int c4 = sl * 4 + 32 * k;
         float4 v = make_float4(acc[a][k][0] * inv, acc[a][k][1] * inv, acc[a][k][2] * inv, acc[a][k][3] * inv);
-        if (c4 < D) st4(kappa + ent * D + c4, v);
-        else st4(nu + ent * D + (c4 - D), v);
+        if (c4 < D) {
+          if (live) st_kappa4<T>(sp, ent * D + c4, v);
+          float4 q = ld4(qb + (ip * 2 + a) * LDQ + c4);
+          qk += q.x * kappa_repr<T>(v.x) + q.y * kappa_repr<T>(v.y) + q.z * kappa_repr<T>(v.z) + q.w * kappa_repr<T>(v.w);
+        } else if (live) {
+          st_nu4<T>(sp, ent * D + (c4 - D), v);
+        }
+      }
+      qk += __shfl_xor_sync(0xffffffffu, qk, 1); qk += __shfl_xor_sync(0xffffffffu, qk, 2); qk += __shfl_xor_sync(0xffffffffu, qk, 4);
+      if (sl == 0 && live) {
+        const float m_ = some ? M[a] + logf(s[a]) : -INFINITY;
+        sp.mu[ent] = m_;
+        sp.beta[ent] = some ? m_ - qk : -INFINITY;
       }
     }
   }
@@ -171,8 +184,7 @@ static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const i
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid(d.Ck, cdiv(d.Cq, kSumI), d.B * d.Hq);
   prof_mark("k_summarize", st);
-  k_summarize<T, D><<<grid, kSumThreads, smem, st>>>(d, Kp, Vp, off_k, qbar, (float*)(base + L.mu),
-                                                    (float*)(base + L.kappa), (float*)(base + L.nu));
+  k_summarize<T, D><<<grid, kSumThreads, smem, st>>>(d, Kp, Vp, off_k, qbar, summ_ptrs(L, base));
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }

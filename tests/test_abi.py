@@ -35,9 +35,10 @@ def test_workspace_sizes_and_layout(mb):
     p = mb.make_params(B=1, Hq=16, Hkv=16, N=65536, D=128, Cq=256, Ck=1024, m=32)
     sizes = mb.muse_workspace_bytes(p)
     ent = 16 * 7 * 256 * 1024
-    assert sizes[4] >= ent * (2 * 128 + 1) * 4 + 2 * 16 * 65536 * 128 * 2
+    assert sizes[4] >= ent * (3 * 128 * 2 + 8) + 2 * 16 * 65536 * 128 * 2
     off = mb.muse_summaries_layout(p)
-    assert off[0] == 0 and off[1] >= ent * 4 and off[2] - off[1] >= ent * 128 * 4 and all(o % 256 == 0 for o in off)
+    assert off[0] == 0 and off[1] >= ent * 4 and off[3] - off[2] >= ent * 128 * 2 and all(o % 256 == 0 for o in off)
+    assert len(off) == 7 and list(off) == sorted(off)
     assert all(s % 256 == 0 for s in sizes)
 
 

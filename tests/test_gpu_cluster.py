@@ -16,7 +16,8 @@ pytestmark = pytest.mark.gpu
 CASES = {
     "tiny": wl.WORKLOADS["tiny"],
     "gqa_bf16": wl.WORKLOADS["small"].with_(B=2, Hq=4, Hkv=2, N=2000, Cq=16, Ck=40, m=6, components=64),
-    "d128": wl.WORKLOADS["headline"].with_(Hq=2, Hkv=1, N=3072, Cq=24, Ck=96, m=8, components=96),
+    "d128": wl.WORKLOADS["headline"].with_(Hq=2, Hkv=1, N=3072, Cq=24, Ck=128, m=8, components=96),
+    "d128_wide": wl.WORKLOADS["headline"].with_(name="headline_wide", Hq=1, Hkv=1, N=2048, Cq=4, Ck=256, m=16, components=64),
 }
 
 

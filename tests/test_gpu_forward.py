@@ -47,7 +47,8 @@ def test_summaries_match_oracle(name, gain):
     Q, K, V, _ = c.dev()
     _run_summaries(mb, c, p, buf, K, V)
     torch.cuda.synchronize()
-    mu, ka, nu = (to_np(x) for x in buf.summary_planes())
+    mu, beta, ka, nu = (to_np(x) for x in buf.summary_planes())
+    t_nu = 1e-4 if w.dtype == "f32" else tol(w.dtype)     # nu is stored in bf16 in bf16 mode
     for b in range(w.B):
         for h in range(w.Hq):
             g = c.hm[h]
@@ -58,7 +59,9 @@ def test_summaries_match_oracle(name, gain):
             fin = np.isfinite(e_mu)
             assert np.abs(e_mu[fin] - g_mu[fin]).max() <= 1e-4 * max(1.0, np.abs(e_mu[fin]).max())
             assert rel_err(ka[b, h], kah[1:]) <= 1e-4
-            assert rel_err(nu[b, h], nuh[1:]) <= 1e-4
+            assert rel_err(nu[b, h], nuh[1:]) <= t_nu
+            e_beta = e_mu - c.sigma * np.einsum("id,bijd->bij", c.qbar32[b, h].astype(np.float64), kah[1:])
+            assert np.abs(e_beta[fin] - beta[b, h][fin]).max() <= 1e-4 * max(1.0, np.abs(e_beta[fin]).max())
 
 
 def _forward_parity(w, gain, sel_mode=0, causal=True):
