@@ -131,7 +131,7 @@ MUSE_API int muse_summarize(const muse_params_t* p, const void* K, const void* V
  *   sel_in   in   [B,Hq,N,m] clusters to retrieve (-1 = none) or NULL to select here
  *   O        out  [B,Hq,N,D] dtype
  *   LSE      out  [B,Hq,N] fp32 log of the merged normaliser
- *   sel_out  out  [B,Hq,N,m] retrieved clusters, best first, padded with -1 (may be NULL) */
+ *   sel_out  out  [B,Hq,N,m] retrieved clusters in no particular order, padded with -1 (may be NULL) */
 MUSE_API int muse_attn_fwd(const muse_params_t* p, const void* Q, const void* K, const void* V,
                   const int32_t* assign_q, const float* qbar,
                   const int32_t* off_k, const int32_t* perm_k, const void* summaries,

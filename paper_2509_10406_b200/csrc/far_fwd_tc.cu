@@ -26,7 +26,9 @@ constexpr int kFarTcCols = 512;
 
 struct FarBars { uint64_t fullA[2], emptyA[2], fullD[4], emptyD[4], done; };
 
-__global__ void __launch_bounds__(128)
+constexpr int kFarTcThreads = 512;      // 16 warps: the per-query selection (phase C) is the long pole
+
+__global__ void __launch_bounds__(kFarTcThreads, 1)
 k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_constant__ CUtensorMap tm_klo,
              const __grid_constant__ CUtensorMap tm_nu, const bf16* __restrict__ Q, const int32_t* __restrict__ off_q,
              const int32_t* __restrict__ perm_q, const float* __restrict__ mu, const float* __restrict__ beta,
@@ -88,9 +90,12 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 
   for (int r0 = p0; r0 < p1 && ok; r0 += kFR) {
     const int n = min(kFR, p1 - r0);
+#ifdef MUSE_PHASE_CLOCKS
+    long long ck0 = clock64(), ck1 = 0, ck2 = 0, ck3 = 0, ck4 = 0;
+#endif
     if (tid < kFR) rows[tid] = tid < n ? pm[r0 + tid] : -1;
     // query rows -> K-major swizzled tile [32][128] bf16 (2 blocks of [32][128 B])
-    for (int e = tid; e < kFR * (kFD / 8); e += 128) {
+    for (int e = tid; e < kFR * (kFD / 8); e += kFarTcThreads) {
       const int r = e >> 4, ck = e & 15, kb = ck >> 3, c = ck & 7;
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
       if (r < n) v = reinterpret_cast<const uint4*>(Qp + (size_t)pm[r0 + r] * kFD)[ck];
@@ -130,24 +135,34 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       }
       tc::mma_commit(&bars.done);
     }
+    __syncwarp();     // lanes 1..31 of warp 0 park here instead of spinning beside the issuing lane
     if (!tc::mbar_wait(&bars.done, done_ph)) ok = false;
     done_ph ^= 1;
     tc::fence_after_sync();
+#ifdef MUSE_PHASE_CLOCKS
+    ck1 = clock64();
+#endif
     // ---- B: TMEM -> sc[r][j]
-    for (int jt = 0; jt < NJ; ++jt) {
+    for (int jt = warp >> 2; jt < NJ; jt += kFarTcThreads / 128) {
       float v[32];
-      tc::tmem_ld32(tbase + ((uint32_t)(warp * 32) << 16) + jt * kFR, v);
-      const int j = jt * kFJ + tid;
+      tc::tmem_ld32(tbase + ((uint32_t)((warp & 3) * 32) << 16) + jt * kFR, v);
+      const int j = jt * kFJ + (tid & 127);
       const float b = bep[j];
 #pragma unroll
       for (int r = 0; r < kFR; ++r) sc[r * Ck + j] = b == -INFINITY ? -INFINITY : fmaf(v[r], dm.sigma, b);
     }
     tc::fence_before_sync();
     __syncthreads();
+#ifdef MUSE_PHASE_CLOCKS
+    ck2 = clock64();
+#endif
     // ---- C: selection + softmax of the far set; P (bf16) -> R1 as a K-major operand [32][Ck]
-    for (int r = warp; r < kFR; r += 4) {
+    for (int r = warp; r < kFR; r += kFarTcThreads / 32) {
       float* s = sc + r * Ck;
       float sum = 0.f, mx = -INFINITY;
+#ifdef MUSE_PHASE_CLOCKS
+      long long cc0 = clock64(), cc1 = 0, cc2 = 0;
+#endif
       if (r < n) {
         const int t = rows[r];
         int32_t* so = sel_out + ((size_t)pq * dm.N + t) * m;
@@ -156,29 +171,65 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
           for (int k = lane; k < m; k += 32) { int c = si[k]; so[k] = c; if (c >= 0 && c < Ck) s[c] = -INFINITY; }
         } else if (dm.sel_mode == MUSE_SEL_PER_QCLUSTER) {
           for (int k = lane; k < m; k += 32) { int c = selq[k]; so[k] = c; if (c >= 0) s[c] = -INFINITY; }
-        } else {
-          float lv = -INFINITY; int li = 0x7fffffff;
-          for (int j = lane; j < Ck; j += 32) { float v = s[j]; if (v > lv) { lv = v; li = j; } }
-          for (int k = 0; k < m; ++k) {
-            float bv = lv; int bi = li;
+        } else if (m > 0) {
+          // Top-m by bisection on an order-preserving integer key of the score: find the key T
+          // of the m-th largest with warp ballots (no serial arg-max rounds), take everything
+          // above T and, among ties at T, the lowest cluster indices.
+          const int NK = Ck >> 5;                       // scores per lane (<= 32)
+          uint32_t key[32];
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-              float ov = __shfl_xor_sync(0xffffffffu, bv, o); int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-              if (ov > bv || (ov == bv && oi < bi)) { bv = ov; bi = oi; }
-            }
-            const bool any = bv != -INFINITY;
-            if (lane == 0) so[k] = any ? bi : -1;
-            if (any && (bi & 31) == lane) {
-              s[bi] = -INFINITY;
-              lv = -INFINITY; li = 0x7fffffff;
-              for (int j = lane; j < Ck; j += 32) { float v = s[j]; if (v > lv) { lv = v; li = j; } }
+          for (int k = 0; k < 32; ++k) {
+            const uint32_t b = __float_as_uint(k < NK ? s[lane + 32 * k] : -INFINITY);
+            key[k] = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+          }
+          const uint32_t kFinite = 0x00800000u;         // smallest key above key(-inf) = 0x007fffff
+          auto count_ge = [&](uint32_t thr) {          // lane-local count, then one warp reduction
+            int c = 0;
+#pragma unroll
+            for (int k = 0; k < 32; ++k) c += key[k] >= thr ? 1 : 0;
+            return (int)__reduce_add_sync(0xffffffffu, (unsigned)c);
+          };
+          uint32_t T = kFinite;
+          if (count_ge(kFinite) > m) {
+            // the leading bits shared by the largest and the smallest finite key need no search
+            uint32_t kmx = 0u, kmn = 0xffffffffu;
+#pragma unroll
+            for (int k = 0; k < 32; ++k) { kmx = max(kmx, key[k]); kmn = min(kmn, key[k] >= kFinite ? key[k] : 0xffffffffu); }
+            kmx = __reduce_max_sync(0xffffffffu, kmx);
+            kmn = __reduce_min_sync(0xffffffffu, kmn);
+            const int shared = __clz((int)(kmx ^ kmn));            // 32 if all finite keys are equal
+            T = shared >= 32 ? kmx : (kmx & ~(0xffffffffu >> shared));
+            for (int bit = 31 - shared; bit >= 0; --bit) {
+              const uint32_t cand = T | (1u << bit);
+              const int c = count_ge(cand);
+              if (c >= m) { T = cand; if (c == m) break; }
             }
           }
+          const int need = m - count_ge(T + 1);         // ties at T to take (all of them if T == kFinite)
+          const uint32_t lt = (1u << lane) - 1u;
+          int base = 0, ties_seen = 0;
+#pragma unroll
+          for (int k = 0; k < 32; ++k) {
+            if (k < NK) {
+              const bool tie = key[k] == T && T != kFinite ? true : false;
+              const bool gt = T == kFinite ? key[k] >= T : key[k] > T;
+              const uint32_t mt = __ballot_sync(0xffffffffu, tie);
+              const bool take = gt || (tie && ties_seen + __popc(mt & lt) < need);
+              ties_seen += __popc(mt);
+              const uint32_t ms = __ballot_sync(0xffffffffu, take);
+              if (take) { so[base + __popc(ms & lt)] = lane + 32 * k; s[lane + 32 * k] = -INFINITY; }
+              base += __popc(ms);
+            }
+          }
+          for (int k = base + lane; k < m; k += 32) so[k] = -1;
         }
         __syncwarp();
         for (int j = lane; j < Ck; j += 32) mx = fmaxf(mx, s[j]);
         mx = warp_max(mx);
       }
+#ifdef MUSE_PHASE_CLOCKS
+      cc1 = clock64();
+#endif
       // probabilities, 8 consecutive clusters (one 16-byte chunk) per lane and step
       for (int q = lane; q < Ck / 8; q += 32) {
         uint32_t w[4];
@@ -192,6 +243,10 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
         }
         *reinterpret_cast<uint4*>(R1 + (q >> 3) * (kFR * 128) + tc::sw128_off(r, q & 7)) = make_uint4(w[0], w[1], w[2], w[3]);
       }
+#ifdef MUSE_PHASE_CLOCKS
+      cc2 = clock64();
+      if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 3 && blockIdx.z == 0 && r0 == p0 && r == 0) { status[13] = (int)(cc1 - cc0); status[14] = (int)(cc2 - cc1); }
+#endif
       sum = warp_sum(sum);
       if (lane == 0) {
         rinv[r] = sum > 0.f ? 1.f / sum : 0.f;
@@ -201,6 +256,9 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     tc::fence_async_smem();
     tc::fence_before_sync();
     __syncthreads();
+#ifdef MUSE_PHASE_CLOCKS
+    ck3 = clock64();
+#endif
     // ---- D: out^T = nu^T P^T, nu tiles through an nsD-stage TMA ring in the score region;
     //         loads run nsD - 1 tiles ahead of the MMAs
     if (tid == 0 && ok) {
@@ -235,11 +293,19 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       }
       tc::mma_commit(&bars.done);
     }
+    __syncwarp();
     if (!tc::mbar_wait(&bars.done, done_ph)) ok = false;
     done_ph ^= 1;
     tc::fence_after_sync();
+#ifdef MUSE_PHASE_CLOCKS
+    ck4 = clock64();
+    if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 3 && blockIdx.z == 0 && r0 == p0) {
+      status[8] = (int)(ck1 - ck0); status[9] = (int)(ck2 - ck1); status[10] = (int)(ck3 - ck2); status[11] = (int)(ck4 - ck3);
+      status[12] = n;
+    }
+#endif
     // ---- E: thread = output dim d
-    {
+    if (warp < 4) {
       float v[32];
       tc::tmem_ld32(tbase + ((uint32_t)(warp * 32) << 16) + 256, v);
       if (ok) {
@@ -276,7 +342,7 @@ int far_fwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const int32_t* 
   const size_t smem = (size_t)kR1Bytes + r2_bytes + kFR * kFD * 2 + 1024;
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_fwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prof_mark("k_far_fwd_tc", st);
-  k_far_fwd_tc<<<dim3(d.Cq, d.SB, d.B * d.Hq), 128, smem, st>>>(d, khi, klo, nu, (const bf16*)Q, off_q, perm_q, sp.mu, sp.beta,
+  k_far_fwd_tc<<<dim3(d.Cq, d.SB, d.B * d.Hq), kFarTcThreads, smem, st>>>(d, khi, klo, nu, (const bf16*)Q, off_q, perm_q, sp.mu, sp.beta,
                                                                sel_in, sel_out, o_far, lse_far, r2_bytes, nsD, status);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
