@@ -5,6 +5,7 @@
 // (Appendix "Aggregation Weight Gradient Flow").
 #include "common.cuh"
 #include "flash_core.cuh"
+#include <cstdlib>
 
 namespace muse {
 
@@ -460,11 +461,11 @@ k_far_bwd(Dims dm, const T* __restrict__ Q, const T* __restrict__ dO, const floa
 // and w_iu = exp(sigma qbar_i . k_u - mu_ij(b')) <= 1:
 //   dK_u += sum_i w_iu [ GU_i + agg (GS_i + GU_i . k_u + GW_i . v_u) sigma qbar_i ],  dV_u += sum_i w_iu GW_i.
 // ---------------------------------------------------------------------------------------------
-template <class T, int D>
+template <class T, int D, class GT>     // GT: storage type of the summary gradients (float or bf16)
 __global__ void __launch_bounds__(kFlashThreads)
 k_summ_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const int32_t* __restrict__ off_k,
            const int32_t* __restrict__ off_q, const float* __restrict__ qbar, const float* __restrict__ mu,
-           const float* __restrict__ dkappa, const float* __restrict__ dnu, const float* __restrict__ dS,
+           const GT* __restrict__ dkappa, const GT* __restrict__ dnu, const float* __restrict__ dS,
            float* __restrict__ dK_perm, float* __restrict__ dV_perm) {
   constexpr int LD = D + 4;
   extern __shared__ __align__(16) unsigned char smraw[];
@@ -637,6 +638,11 @@ int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, con
                const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, float* dq_part,
                float* dK_perm, float* dV_perm, int* status, cudaStream_t st);
 
+bool far_bwd_tc_supported(const Dims& d, int dtype);
+int far_bwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const void* dO, const float* qbar, const float* LSE,
+               const float* delta, const int32_t* off_q, const int32_t* perm_q, const int32_t* sel, float* dQacc,
+               void* dkappa, void* dnu, float* dS, int* status, cudaStream_t st);
+
 struct BwdWs {
   int32_t *status, *off_q, *perm_q, *sort_scratch, *ret_scratch;
   float *delta, *dQacc, *dq_part, *dK_orig, *dV_orig, *dK_perm, *dV_perm, *dkappa, *dnu, *dS;
@@ -726,17 +732,31 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
       }
       use_ret = 1;
     }
+    const bool far_tc = far_bwd_tc_supported(d, dtype) && getenv("MUSE_FAR_SIMT") == nullptr;
     const size_t fsm = (size_t)(4 * kTile * (D + 4) + kTile * kLDP) * sizeof(float) + (size_t)kTile * cdiv(d.Ck, 32) * sizeof(uint32_t);
+    if (far_tc) {
+      rc = far_bwd_tc(d, sp, Q, dO, qbar, LSE, w.delta, w.off_q, w.perm_q, sel, w.dQacc, w.dkappa, w.dnu, w.dS, w.status, st);
+      if (rc != MUSE_OK) return rc;
+    } else {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fsm));
     prof_mark("k_far_bwd", st);
     k_far_bwd<T, D><<<dim3(d.Cq, d.SB, pq), kFlashThreads, fsm, st>>>(d, Q, dO, qbar, LSE, w.delta, w.off_q, w.perm_q, sel, sp,
                                                                     w.dQacc, w.dkappa, w.dnu, w.dS);
     MUSE_LAUNCH_OK();
+    }
     const size_t ssm = (size_t)(5 * kTile * (D + 4) + kTile * kLDP) * sizeof(float);
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
-    prof_mark("k_summ_bwd", st);
-    k_summ_bwd<T, D><<<dim3(d.Ck, pq), kFlashThreads, ssm, st>>>(d, Kp, Vp, off_k, w.off_q, qbar, mu, w.dkappa, w.dnu, w.dS,
-                                                               w.dK_perm, w.dV_perm);
+    if (far_tc) {
+      typedef __nv_bfloat16 GB;
+      MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd<T, D, GB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
+      prof_mark("k_summ_bwd", st);
+      k_summ_bwd<T, D, GB><<<dim3(d.Ck, pq), kFlashThreads, ssm, st>>>(d, Kp, Vp, off_k, w.off_q, qbar, mu, (const GB*)w.dkappa,
+                                                                     (const GB*)w.dnu, w.dS, w.dK_perm, w.dV_perm);
+    } else {
+      MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd<T, D, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
+      prof_mark("k_summ_bwd", st);
+      k_summ_bwd<T, D, float><<<dim3(d.Ck, pq), kFlashThreads, ssm, st>>>(d, Kp, Vp, off_k, w.off_q, qbar, mu, w.dkappa, w.dnu, w.dS,
+                                                                        w.dK_perm, w.dV_perm);
+    }
     MUSE_LAUNCH_OK();
   }
   prof_mark("k_final_dq", st);

@@ -1,0 +1,276 @@
+// Far-field backward on the tensor cores (bf16 mode, D = 128, Ck a multiple of 128, <= 1024).
+// One CTA per (query cluster i, plane, head) segment.  Clusters sit on the MMA M side (128 per
+// tile, one TMEM lane each), the segment's queries on the N side (64 per pass, two passes
+// resident).  Per cluster tile, with L the merged log-sum-exp and delta = dO.O:
+//   S^T   = (kappa_hi + kappa_lo) Q^T,  dPnu^T = nu dO^T                      (tcgen05, TMA-fed tiles)
+//   p     = exp(sigma S + beta - L) on the far set,  g = p (dPnu - delta)      (one thread per cluster)
+//   dnu  += p dO,   dkappa_raw += g Q,   dq^T += kappa^T g                     (tcgen05)
+//   dkappa = sigma (dkappa_raw - (sum_r g) qbar_i),   dS = sum_r g - dkappa.kappa - dnu.nu
+// dkappa and dnu are stored as bf16 rows for the key-side pass, dS as fp32.
+#include <cuda.h>
+#include "common.cuh"
+#include "tc05.cuh"
+
+namespace muse {
+
+typedef __nv_bfloat16 bf16;
+int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
+
+namespace fb {
+constexpr int D = 128, TJ = 128, NR = 64, NP = 2, THREADS = 256;
+constexpr int kTile = TJ * D * 2;                 // 32 KB operand tile [128][128] bf16
+constexpr int kRows = NR * D * 2;                 // 16 KB tile of 64 query rows
+constexpr int oHi = 0, oLo = oHi + kTile, oNu = oLo + kTile;
+constexpr int oQ = oNu + kTile, oDO = oQ + NP * kRows;
+constexpr int oPt = oDO + NP * kRows, oGt = oPt + TJ * NR * 2;
+constexpr int oMask = oGt + TJ * NR * 2;          // [NP*NR rows][Ck/32] words follow
+constexpr uint32_t cS = 0, cDP = 64, cDNU = 128, cDKA = 256, cDQ = 384;   // TMEM columns
+constexpr float kLog2e = 1.4426950408889634f;
+}  // namespace fb
+
+__global__ void __launch_bounds__(fb::THREADS, 1)
+k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_constant__ CUtensorMap tm_klo,
+             const __grid_constant__ CUtensorMap tm_nu, const bf16* __restrict__ Q, const bf16* __restrict__ dO,
+             const float* __restrict__ qbar, const float* __restrict__ LSE, const float* __restrict__ delta,
+             const int32_t* __restrict__ off_q, const int32_t* __restrict__ perm_q, const int32_t* __restrict__ sel,
+             const float* __restrict__ beta, float* __restrict__ dQacc, bf16* __restrict__ dkappa,
+             bf16* __restrict__ dnu, float* __restrict__ dS, int* __restrict__ status) {
+  using namespace fb;
+  extern __shared__ __align__(1024) unsigned char sm_raw[];
+  __shared__ uint64_t bar_full, bar1, bar2;
+  __shared__ uint32_t tbase_s;
+  __shared__ int32_t rows[NP * NR];
+  __shared__ float Ls[NP * NR], ds[NP * NR], qb[D], part[2][TJ], dots[2][TJ];
+  const int i = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z;
+  const int blk = dm.causal ? pl + 1 : 0, Ck = dm.Ck, NJ = Ck / TJ, MW = Ck >> 5, m = dm.m;
+  const int tid = threadIdx.x, warp = tid >> 5, wg = tid >> 7, L = tid & 127;
+  const int32_t* oq = off_q + (size_t)pq * (dm.S * dm.Cq + 1) + (size_t)blk * dm.Cq + i;
+  const int p0 = oq[0], p1 = oq[1];
+  if (p0 >= p1) return;
+  unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
+  uint32_t* smask = reinterpret_cast<uint32_t*>(sm + oMask);
+  const size_t ent0 = (((size_t)pq * dm.SB + pl) * dm.Cq + i) * Ck;
+  const bf16* Qp = Q + (size_t)pq * dm.N * D;
+  const bf16* dOp = dO + (size_t)pq * dm.N * D;
+  const int32_t* pm = perm_q + (size_t)pq * dm.N;
+
+  if (warp == 0) tc::tmem_alloc(&tbase_s, 512);
+  if (tid == 0) { tc::mbar_init(&bar_full, 1); tc::mbar_init(&bar1, 1); tc::mbar_init(&bar2, 1); tc::mbar_init_fence(); }
+  if (tid < D) qb[tid] = qbar[((size_t)pq * dm.Cq + i) * D + tid];
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tbase = tbase_s, tlane = tbase + ((uint32_t)((warp & 3) * 32) << 16);
+  uint32_t ph_full = 0, ph1 = 0, ph2 = 0;
+  bool ok = true;
+  const uint32_t aHi = tc::smem_u32(sm + oHi), aLo = tc::smem_u32(sm + oLo), aNu = tc::smem_u32(sm + oNu),
+                 aPt = tc::smem_u32(sm + oPt), aGt = tc::smem_u32(sm + oGt);
+
+  for (int s0 = p0; s0 < p1 && ok; s0 += NP * NR) {        // super-pass: up to 128 rows
+    const int ns = min(NP * NR, p1 - s0), np = (ns + NR - 1) / NR;
+    __syncthreads();
+    if (tid < NP * NR) {
+      const int t = tid < ns ? pm[s0 + tid] : -1;
+      rows[tid] = t;
+      Ls[tid] = t >= 0 ? LSE[(size_t)pq * dm.N + t] * kLog2e : 0.f;
+      ds[tid] = t >= 0 ? delta[(size_t)pq * dm.N + t] : 0.f;
+    }
+    for (int e = tid; e < NP * NR * MW; e += THREADS) smask[e] = 0u;
+    __syncthreads();
+    for (int e = tid; e < NP * NR * (D / 8); e += THREADS) {
+      const int r = e >> 4, ck = e & 15, kb = ck >> 3, c = ck & 7, p = r / NR, rr = r % NR;
+      uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+      if (r < ns) {
+        a = reinterpret_cast<const uint4*>(Qp + (size_t)rows[r] * D)[ck];
+        b = reinterpret_cast<const uint4*>(dOp + (size_t)rows[r] * D)[ck];
+      }
+      *reinterpret_cast<uint4*>(sm + oQ + p * kRows + kb * NR * 128 + tc::sw128_off(rr, c)) = a;
+      *reinterpret_cast<uint4*>(sm + oDO + p * kRows + kb * NR * 128 + tc::sw128_off(rr, c)) = b;
+    }
+    for (int e = tid; e < ns * m; e += THREADS) {
+      const int r = e / m, k = e % m;
+      const int c = sel[((size_t)pq * dm.N + rows[r]) * m + k];
+      if (c >= 0 && c < Ck) atomicOr(&smask[r * MW + (c >> 5)], 1u << (c & 31));
+    }
+    tc::fence_async_smem();
+    __syncthreads();
+
+    for (int jt = 0; jt < NJ && ok; ++jt) {
+      const int j = jt * TJ + L;
+      if (tid == 0) {
+        tc::mbar_expect_tx(&bar_full, 3 * kTile);
+        const int row = (int)(ent0 + (size_t)jt * TJ);
+        tc::tma_load_2d(sm + oHi, &tm_khi, 0, row, &bar_full); tc::tma_load_2d(sm + oHi + TJ * 128, &tm_khi, 64, row, &bar_full);
+        tc::tma_load_2d(sm + oLo, &tm_klo, 0, row, &bar_full); tc::tma_load_2d(sm + oLo + TJ * 128, &tm_klo, 64, row, &bar_full);
+        tc::tma_load_2d(sm + oNu, &tm_nu, 0, row, &bar_full); tc::tma_load_2d(sm + oNu + TJ * 128, &tm_nu, 64, row, &bar_full);
+      }
+      const float bj = beta[ent0 + j];
+      float gsum = 0.f;
+      for (int p = 0; p < np && ok; ++p) {
+        const uint32_t aQ = tc::smem_u32(sm + oQ + p * kRows), aDO = tc::smem_u32(sm + oDO + p * kRows);
+        if (tid == 0) {
+          if (p == 0) { if (!tc::mbar_wait(&bar_full, ph_full)) ok = false; }
+          tc::fence_after_sync();
+          const uint32_t idesc = tc::idesc_bf16(TJ, NR, 0, 0);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks)
+            tc::mma_bf16_ss(tbase + cS, tc::smem_desc_sw128(aHi + (ks / 4) * TJ * 128 + (ks % 4) * 32, 16, 1024),
+                            tc::smem_desc_sw128(aQ + (ks / 4) * NR * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks)
+            tc::mma_bf16_ss(tbase + cS, tc::smem_desc_sw128(aLo + (ks / 4) * TJ * 128 + (ks % 4) * 32, 16, 1024),
+                            tc::smem_desc_sw128(aQ + (ks / 4) * NR * 128 + (ks % 4) * 32, 16, 1024), idesc, 1);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks)
+            tc::mma_bf16_ss(tbase + cDP, tc::smem_desc_sw128(aNu + (ks / 4) * TJ * 128 + (ks % 4) * 32, 16, 1024),
+                            tc::smem_desc_sw128(aDO + (ks / 4) * NR * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
+          tc::mma_commit(&bar1);
+        }
+        __syncwarp();
+        if (!tc::mbar_wait(&bar1, ph1)) ok = false;
+        ph1 ^= 1;
+        tc::fence_after_sync();
+        {
+          float s[32], dp[32];
+          tc::tmem_ld32(tlane + cS + 32 * wg, s);
+          tc::tmem_ld32(tlane + cDP + 32 * wg, dp);
+          uint32_t pw[16], gw[16];
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            float pv[2], gv[2];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int r = p * NR + 32 * wg + c + h;
+              const bool far = bj != -INFINITY && r < ns && !((smask[r * MW + (j >> 5)] >> (j & 31)) & 1u);
+              pv[h] = far ? exp2f(fmaf(s[c + h], dm.sigma, bj) * kLog2e - Ls[r]) : 0.f;
+              gv[h] = pv[h] * (dp[c + h] - ds[r]);
+              gsum += gv[h];
+            }
+            __nv_bfloat162 a = __floats2bfloat162_rn(pv[0], pv[1]), b = __floats2bfloat162_rn(gv[0], gv[1]);
+            pw[c >> 1] = *reinterpret_cast<uint32_t*>(&a);
+            gw[c >> 1] = *reinterpret_cast<uint32_t*>(&b);
+          }
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {
+            *reinterpret_cast<uint4*>(sm + oPt + tc::sw128_off(L, 4 * wg + ch)) = make_uint4(pw[4 * ch], pw[4 * ch + 1], pw[4 * ch + 2], pw[4 * ch + 3]);
+            *reinterpret_cast<uint4*>(sm + oGt + tc::sw128_off(L, 4 * wg + ch)) = make_uint4(gw[4 * ch], gw[4 * ch + 1], gw[4 * ch + 2], gw[4 * ch + 3]);
+          }
+        }
+        tc::fence_async_smem();
+        tc::fence_before_sync();
+        __syncthreads();
+        if (tid == 0) {
+          tc::fence_after_sync();
+          const uint32_t id_row = tc::idesc_bf16(TJ, D, 0, 1);      // A K-major (P / G), B = query rows, MN-major
+          const uint32_t id_dq = tc::idesc_bf16(D, NR, 1, 1);       // A = kappa tile MN-major, B = G MN-major
+#pragma unroll
+          for (int ks = 0; ks < NR / 16; ++ks)
+            tc::mma_bf16_ss(tbase + cDNU, tc::smem_desc_sw128(aPt + ks * 32, 16, 1024),
+                            tc::smem_desc_sw128(aDO + ks * 16 * 128, NR * 128, 1024), id_row, !(p == 0 && ks == 0));
+#pragma unroll
+          for (int ks = 0; ks < NR / 16; ++ks)
+            tc::mma_bf16_ss(tbase + cDKA, tc::smem_desc_sw128(aGt + ks * 32, 16, 1024),
+                            tc::smem_desc_sw128(aQ + ks * 16 * 128, NR * 128, 1024), id_row, !(p == 0 && ks == 0));
+#pragma unroll
+          for (int ks = 0; ks < TJ / 16; ++ks)
+            tc::mma_bf16_ss(tbase + cDQ + p * NR, tc::smem_desc_sw128(aHi + ks * 16 * 128, TJ * 128, 1024),
+                            tc::smem_desc_sw128(aGt + ks * 16 * 128, TJ * 128, 1024), id_dq, !(jt == 0 && ks == 0));
+#pragma unroll
+          for (int ks = 0; ks < TJ / 16; ++ks)
+            tc::mma_bf16_ss(tbase + cDQ + p * NR, tc::smem_desc_sw128(aLo + ks * 16 * 128, TJ * 128, 1024),
+                            tc::smem_desc_sw128(aGt + ks * 16 * 128, TJ * 128, 1024), id_dq, 1);
+          tc::mma_commit(&bar2);
+        }
+        __syncwarp();
+        if (!tc::mbar_wait(&bar2, ph2)) ok = false;
+        ph2 ^= 1;
+        tc::fence_after_sync();
+      }
+      ph_full ^= 1;
+      // ---- tile read-out: warpgroup 0 -> dnu, warpgroup 1 -> dkappa; both need sum_r g
+      part[wg][L] = gsum;
+      __syncthreads();
+      const float gtot = part[0][L] + part[1][L];
+      float dot = 0.f;
+      bf16* dst = (wg == 0 ? dnu : dkappa) + (ent0 + j) * D;
+#pragma unroll
+      for (int d0 = 0; d0 < D; d0 += 32) {
+        float v[32];
+        tc::tmem_ld32(tlane + (wg == 0 ? cDNU : cDKA) + d0, v);
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          const int d = d0 + 8 * ch, kb = d >> 6, c = (d & 63) >> 3;
+          const uint32_t off = kb * TJ * 128 + tc::sw128_off(L, c);
+          float x[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) x[e] = wg == 0 ? v[8 * ch + e] : dm.sigma * (v[8 * ch + e] - gtot * qb[d + e]);
+          uint4 ra = *reinterpret_cast<const uint4*>(sm + (wg == 0 ? oNu : oHi) + off);
+          const bf16* ha = reinterpret_cast<const bf16*>(&ra);
+          if (wg == 0) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) dot = fmaf(x[e], __bfloat162float(ha[e]), dot);
+          } else {
+            uint4 rb = *reinterpret_cast<const uint4*>(sm + oLo + off);
+            const bf16* hb = reinterpret_cast<const bf16*>(&rb);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) dot = fmaf(x[e], __bfloat162float(ha[e]) + __bfloat162float(hb[e]), dot);
+          }
+          uint32_t w[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) { __nv_bfloat162 b2 = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]); w[e] = *reinterpret_cast<uint32_t*>(&b2); }
+          if (ok) *reinterpret_cast<uint4*>(dst + d) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      dots[wg][L] = dot;
+      tc::fence_async_smem();          // generic reads of the tiles are ordered before the next TMA writes
+      tc::fence_before_sync();
+      __syncthreads();
+      if (wg == 0 && ok) dS[ent0 + j] = gtot - dots[0][L] - dots[1][L];
+    }
+    // ---- dq: warpgroup p reads pass p (thread = output dim), adds into the fp32 accumulator
+    for (int p = wg; p < np; p += 2) {
+#pragma unroll
+      for (int c0 = 0; c0 < NR; c0 += 32) {
+        float v[32];
+        tc::tmem_ld32(tlane + cDQ + p * NR + c0, v);
+        if (ok) {
+#pragma unroll
+          for (int r = 0; r < 32; ++r) {
+            const int rr = p * NR + c0 + r;
+            if (rr < ns) dQacc[((size_t)pq * dm.N + rows[rr]) * D + L] += dm.sigma * v[r];
+          }
+        }
+      }
+    }
+    tc::fence_before_sync();
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tbase, 512);
+  if (!ok && tid == 0) atomicExch(status, 4);
+}
+
+bool far_bwd_tc_supported(const Dims& d, int dtype) {
+  return dtype == MUSE_BF16 && d.D == fb::D && d.Ck % fb::TJ == 0 && d.Ck <= 1024;
+}
+
+int far_bwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const void* dO, const float* qbar, const float* LSE,
+               const float* delta, const int32_t* off_q, const int32_t* perm_q, const int32_t* sel, float* dQacc,
+               void* dkappa, void* dnu, float* dS, int* status, cudaStream_t st) {
+  const uint64_t ent = (uint64_t)d.B * d.Hq * d.SB * d.Cq * d.Ck;
+  CUtensorMap khi, klo, nu;
+  int rc = make_tmap_bf16_rows(&khi, sp.khi, ent, fb::D, fb::TJ);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&klo, sp.klo, ent, fb::D, fb::TJ);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&nu, sp.nu, ent, fb::D, fb::TJ);
+  if (rc != MUSE_OK) return rc;
+  const size_t smem = (size_t)fb::oMask + (size_t)fb::NP * fb::NR * (d.Ck / 32) * 4 + 1024;
+  MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_bwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  prof_mark("k_far_bwd_tc", st);
+  k_far_bwd_tc<<<dim3(d.Cq, d.SB, d.B * d.Hq), fb::THREADS, smem, st>>>(
+      d, khi, klo, nu, (const bf16*)Q, (const bf16*)dO, qbar, LSE, delta, off_q, perm_q, sel, sp.beta, dQacc, (bf16*)dkappa,
+      (bf16*)dnu, dS, status);
+  MUSE_LAUNCH_OK();
+  return MUSE_OK;
+}
+
+}  // namespace muse
