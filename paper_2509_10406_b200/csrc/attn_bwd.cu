@@ -643,6 +643,11 @@ int far_bwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const void* dO,
                const float* delta, const int32_t* off_q, const int32_t* perm_q, const int32_t* sel, float* dQacc,
                void* dkappa, void* dnu, float* dS, int* status, cudaStream_t st);
 
+bool summ_bwd_tc_supported(const Dims& d, int dtype);
+int summ_bwd_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* off_q, const float* qbar,
+                const float* mu, const void* dkappa, const void* dnu, const float* dS, float* dK_perm, float* dV_perm,
+                int* status, cudaStream_t st);
+
 struct BwdWs {
   int32_t *status, *off_q, *perm_q, *sort_scratch, *ret_scratch;
   float *delta, *dQacc, *dq_part, *dK_orig, *dV_orig, *dK_perm, *dV_perm, *dkappa, *dnu, *dS;
@@ -745,7 +750,10 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
     MUSE_LAUNCH_OK();
     }
     const size_t ssm = (size_t)(5 * kTile * (D + 4) + kTile * kLDP) * sizeof(float);
-    if (far_tc) {
+    if (far_tc && summ_bwd_tc_supported(d, dtype) && getenv("MUSE_SUMM_SIMT") == nullptr) {
+      rc = summ_bwd_tc(d, Kp, Vp, off_k, w.off_q, qbar, mu, w.dkappa, w.dnu, w.dS, w.dK_perm, w.dV_perm, w.status, st);
+      if (rc != MUSE_OK) return rc;
+    } else if (far_tc) {
       typedef __nv_bfloat16 GB;
       MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd<T, D, GB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
       prof_mark("k_summ_bwd", st);

@@ -203,7 +203,8 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
           const uint32_t off = kb * TJ * 128 + tc::sw128_off(L, c);
           float x[8];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) x[e] = wg == 0 ? v[8 * ch + e] : dm.sigma * (v[8 * ch + e] - gtot * qb[d + e]);
+          for (int e = 0; e < 8; ++e)      // rounded to the stored bf16 value so that dS matches what the key-side pass reads
+            x[e] = __bfloat162float(__float2bfloat16_rn(wg == 0 ? v[8 * ch + e] : dm.sigma * (v[8 * ch + e] - gtot * qb[d + e])));
           uint4 ra = *reinterpret_cast<const uint4*>(sm + (wg == 0 ? oNu : oHi) + off);
           const bf16* ha = reinterpret_cast<const bf16*>(&ra);
           if (wg == 0) {

@@ -1,0 +1,242 @@
+// Key-side pass of the backward through the accumulated summaries, on the tensor cores
+// (bf16 mode, D = 128, Cq a multiple of 128).  One CTA per (key cluster j, head).  For every
+// plane pl the summary (i, j, pl) was built from the keys u of cluster j in blocks <= pl, with
+// weights w_iu = exp(sigma qbar_i.k_u - mu_ij(pl)) <= 1.  Given the far-field gradients
+// (dkappa, dnu, dS) of that plane:
+//   c_iu  = dS_i + dkappa_i.k_u + dnu_i.v_u
+//   dK_u += sum_i w_iu dkappa_i + [agg_grad] sum_i (w_iu c_iu) (sigma qbar_i),   dV_u += sum_i w_iu dnu_i
+// (the shared-memory qbar tiles already carry the factor sigma)
+// Query clusters sit on the MMA M side for the three D-contractions (one thread per i computes
+// w and w*c) and on the K side for the three i-contractions, whose outputs are transposed
+// ([d][u]) so that the read-out is coalesced over d.  Planes are handled independently.
+#include <cuda.h>
+#include "common.cuh"
+#include "tc05.cuh"
+
+namespace muse {
+
+typedef __nv_bfloat16 bf16;
+
+namespace sb {
+constexpr int D = 128, TI = 128, NU = 64;
+constexpr int kTile = TI * D * 2;              // 32 KB
+constexpr int kKeys = NU * D * 2;              // 16 KB
+constexpr int oQhi = 0, oQlo = oQhi + kTile, oDka = oQlo + kTile, oDnu = oDka + kTile;
+constexpr int oK = oDnu + kTile, oV = oK + kKeys, oW = oV + kKeys, oWc = oW + TI * NU * 2;
+constexpr int total = oWc + TI * NU * 2 + 1024;
+constexpr uint32_t cL = 0, cX1 = 64, cX2 = 128, cDK = 192, cDV = 256;
+}  // namespace sb
+
+// 2-D tensor map over a bf16 matrix with an arbitrary row pitch (bytes), 128B swizzle, box [box_rows][64]
+int make_tmap_bf16_pitched(void* out_map, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows);
+
+__global__ void __launch_bounds__(128, 1)
+k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_constant__ CUtensorMap tm_dnu,
+              const __grid_constant__ CUtensorMap tm_K, const __grid_constant__ CUtensorMap tm_V,
+              const int32_t* __restrict__ off_k, const int32_t* __restrict__ off_q, const float* __restrict__ qbar,
+              const float* __restrict__ mu, const float* __restrict__ dS, float* __restrict__ dK_perm,
+              float* __restrict__ dV_perm, int* __restrict__ status) {
+  using namespace sb;
+  extern __shared__ __align__(1024) unsigned char sm_raw[];
+  __shared__ uint64_t bar_g, bar_kv, bar1, bar2;
+  __shared__ uint32_t tbase_s;
+  const int j = blockIdx.x, pq = blockIdx.y;
+  const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const int32_t* ok_ = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
+  const int32_t* oq = off_q + (size_t)pq * (dm.S * dm.Cq + 1);
+  const int kbeg = ok_[0];
+  if (kbeg >= ok_[dm.SB]) return;                       // no key of this cluster is ever summarised
+  unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
+  if (warp == 0) tc::tmem_alloc(&tbase_s, 512);
+  if (tid == 0) { tc::mbar_init(&bar_g, 1); tc::mbar_init(&bar_kv, 1); tc::mbar_init(&bar1, 1); tc::mbar_init(&bar2, 1); tc::mbar_init_fence(); }
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tbase = tbase_s, tlane = tbase + ((uint32_t)(warp * 32) << 16);
+  uint32_t ph_g = 0, ph_kv = 0, ph1 = 0, ph2 = 0;
+  bool ok = true;
+  const uint32_t aQhi = tc::smem_u32(sm + oQhi), aQlo = tc::smem_u32(sm + oQlo), aDka = tc::smem_u32(sm + oDka),
+                 aDnu = tc::smem_u32(sm + oDnu), aK = tc::smem_u32(sm + oK), aV = tc::smem_u32(sm + oV),
+                 aW = tc::smem_u32(sm + oW), aWc = tc::smem_u32(sm + oWc);
+
+  for (int i0 = 0; i0 < dm.Cq && ok; i0 += TI) {
+    // sigma * qbar tile as bf16 hi + lo (thread = row)
+    __syncthreads();
+    {
+      const int i = i0 + tid;
+      const float* src = qbar + ((size_t)pq * dm.Cq + (i < dm.Cq ? i : 0)) * D;
+#pragma unroll
+      for (int ck = 0; ck < D / 8; ++ck) {
+        uint32_t wh[4], wl[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          float x0 = i < dm.Cq ? src[ck * 8 + 2 * e] * dm.sigma : 0.f, x1 = i < dm.Cq ? src[ck * 8 + 2 * e + 1] * dm.sigma : 0.f;
+          __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+          __nv_bfloat162 ll = __floats2bfloat162_rn(x0 - __low2float(hh), x1 - __high2float(hh));
+          wh[e] = *reinterpret_cast<uint32_t*>(&hh); wl[e] = *reinterpret_cast<uint32_t*>(&ll);
+        }
+        const uint32_t off = (ck >> 3) * TI * 128 + tc::sw128_off(tid, ck & 7);
+        *reinterpret_cast<uint4*>(sm + oQhi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+        *reinterpret_cast<uint4*>(sm + oQlo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
+      }
+    }
+    for (int pl = 0; pl < dm.SB && ok; ++pl) {
+      const int kend = ok_[pl + 1];
+      if (kend <= kbeg) continue;                       // empty prefix: nothing was summarised
+      const int i = i0 + tid, blk = dm.causal ? pl + 1 : 0;
+      const size_t ent = (((size_t)pq * dm.SB + pl) * dm.Cq + (i < dm.Cq ? i : 0)) * dm.Ck + j;
+      const bool live = i < dm.Cq && oq[(size_t)blk * dm.Cq + i + 1] > oq[(size_t)blk * dm.Cq + i];
+      const float mu_i = live ? mu[ent] : 0.f, dS_i = live ? dS[ent] : 0.f;
+      __syncthreads();                                  // previous users of the gradient tiles are done
+      if (tid == 0) {
+        tc::mbar_expect_tx(&bar_g, 2 * kTile);
+        const int row = (int)(((size_t)pq * dm.SB + pl) * dm.Cq + i0), col = j * D;
+        tc::tma_load_2d(sm + oDka, &tm_dka, col, row, &bar_g); tc::tma_load_2d(sm + oDka + TI * 128, &tm_dka, col + 64, row, &bar_g);
+        tc::tma_load_2d(sm + oDnu, &tm_dnu, col, row, &bar_g); tc::tma_load_2d(sm + oDnu + TI * 128, &tm_dnu, col + 64, row, &bar_g);
+      }
+      if (!tc::mbar_wait(&bar_g, ph_g)) ok = false;
+      ph_g ^= 1;
+      // rows of query clusters whose segment is empty were never written: clear them
+      if (!live) {
+#pragma unroll
+        for (int ck = 0; ck < D / 8; ++ck) {
+          const uint32_t off = (ck >> 3) * TI * 128 + tc::sw128_off(tid, ck & 7);
+          *reinterpret_cast<uint4*>(sm + oDka + off) = make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(sm + oDnu + off) = make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+      for (int c0 = kbeg; c0 < kend && ok; c0 += NU) {
+        const int nk = min(NU, kend - c0);
+        tc::fence_async_smem();
+        __syncthreads();                                // K/V tiles and w tiles of the previous chunk are free
+        if (tid == 0) {
+          tc::mbar_expect_tx(&bar_kv, 2 * kKeys);
+          const int row = (int)((size_t)pk * dm.N + c0);
+          tc::tma_load_2d(sm + oK, &tm_K, 0, row, &bar_kv); tc::tma_load_2d(sm + oK + NU * 128, &tm_K, 64, row, &bar_kv);
+          tc::tma_load_2d(sm + oV, &tm_V, 0, row, &bar_kv); tc::tma_load_2d(sm + oV + NU * 128, &tm_V, 64, row, &bar_kv);
+          if (!tc::mbar_wait(&bar_kv, ph_kv)) ok = false;
+          tc::fence_after_sync();
+          const uint32_t idesc = tc::idesc_bf16(TI, NU, 0, 0);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks)
+            tc::mma_bf16_ss(tbase + cL, tc::smem_desc_sw128(aQhi + (ks / 4) * TI * 128 + (ks % 4) * 32, 16, 1024),
+                            tc::smem_desc_sw128(aK + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks)
+            tc::mma_bf16_ss(tbase + cL, tc::smem_desc_sw128(aQlo + (ks / 4) * TI * 128 + (ks % 4) * 32, 16, 1024),
+                            tc::smem_desc_sw128(aK + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, 1);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks)
+            tc::mma_bf16_ss(tbase + cX1, tc::smem_desc_sw128(aDka + (ks / 4) * TI * 128 + (ks % 4) * 32, 16, 1024),
+                            tc::smem_desc_sw128(aK + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks)
+            tc::mma_bf16_ss(tbase + cX2, tc::smem_desc_sw128(aDnu + (ks / 4) * TI * 128 + (ks % 4) * 32, 16, 1024),
+                            tc::smem_desc_sw128(aV + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
+          tc::mma_commit(&bar1);
+        }
+        ph_kv ^= 1;
+        __syncwarp();
+        if (!tc::mbar_wait(&bar1, ph1)) ok = false;
+        ph1 ^= 1;
+        tc::fence_after_sync();
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          float l[32], x1[32], x2[32];
+          tc::tmem_ld32(tlane + cL + 32 * hh, l);
+          tc::tmem_ld32(tlane + cX1 + 32 * hh, x1);
+          tc::tmem_ld32(tlane + cX2 + 32 * hh, x2);
+          uint32_t ww[16], wc[16];
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            float w0 = 0.f, w1 = 0.f, c0_ = 0.f, c1_ = 0.f;
+            if (live && 32 * hh + c < nk) { w0 = __expf(l[c] - mu_i); c0_ = w0 * (dS_i + x1[c] + x2[c]); }
+            if (live && 32 * hh + c + 1 < nk) { w1 = __expf(l[c + 1] - mu_i); c1_ = w1 * (dS_i + x1[c + 1] + x2[c + 1]); }
+            __nv_bfloat162 a = __floats2bfloat162_rn(w0, w1), b = __floats2bfloat162_rn(c0_, c1_);
+            ww[c >> 1] = *reinterpret_cast<uint32_t*>(&a); wc[c >> 1] = *reinterpret_cast<uint32_t*>(&b);
+          }
+#pragma unroll
+          for (int ch = 0; ch < 4; ++ch) {
+            *reinterpret_cast<uint4*>(sm + oW + tc::sw128_off(tid, 4 * hh + ch)) = make_uint4(ww[4 * ch], ww[4 * ch + 1], ww[4 * ch + 2], ww[4 * ch + 3]);
+            *reinterpret_cast<uint4*>(sm + oWc + tc::sw128_off(tid, 4 * hh + ch)) = make_uint4(wc[4 * ch], wc[4 * ch + 1], wc[4 * ch + 2], wc[4 * ch + 3]);
+          }
+        }
+        tc::fence_async_smem();
+        tc::fence_before_sync();
+        __syncthreads();
+        if (tid == 0) {
+          tc::fence_after_sync();
+          const uint32_t idesc = tc::idesc_bf16(D, NU, 1, 1);       // A [i][d] and B [i][u]: both contract over rows
+#pragma unroll
+          for (int ks = 0; ks < TI / 16; ++ks)
+            tc::mma_bf16_ss(tbase + cDK, tc::smem_desc_sw128(aDka + ks * 16 * 128, TI * 128, 1024),
+                            tc::smem_desc_sw128(aW + ks * 16 * 128, TI * 128, 1024), idesc, ks > 0);
+          if (dm.agg_grad) {
+#pragma unroll
+            for (int ks = 0; ks < TI / 16; ++ks)
+              tc::mma_bf16_ss(tbase + cDK, tc::smem_desc_sw128(aQhi + ks * 16 * 128, TI * 128, 1024),
+                              tc::smem_desc_sw128(aWc + ks * 16 * 128, TI * 128, 1024), idesc, 1);
+          }
+#pragma unroll
+          for (int ks = 0; ks < TI / 16; ++ks)
+            tc::mma_bf16_ss(tbase + cDV, tc::smem_desc_sw128(aDnu + ks * 16 * 128, TI * 128, 1024),
+                            tc::smem_desc_sw128(aW + ks * 16 * 128, TI * 128, 1024), idesc, ks > 0);
+          tc::mma_commit(&bar2);
+        }
+        __syncwarp();
+        if (!tc::mbar_wait(&bar2, ph2)) ok = false;
+        ph2 ^= 1;
+        tc::fence_after_sync();
+        // read-out: thread = d, columns = keys of the chunk; add into the fp32 accumulators
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+          float a[32], b[32];
+          tc::tmem_ld32(tlane + cDK + 32 * hh, a);
+          tc::tmem_ld32(tlane + cDV + 32 * hh, b);
+          if (ok) {
+#pragma unroll
+            for (int u = 0; u < 32; ++u) {
+              if (32 * hh + u < nk) {
+                const size_t at = ((size_t)pq * dm.N + c0 + 32 * hh + u) * D + tid;
+                dK_perm[at] += a[u];
+                dV_perm[at] += b[u];
+              }
+            }
+          }
+        }
+        tc::fence_before_sync();
+      }
+    }
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tbase, 512);
+  if (!ok && tid == 0) atomicExch(status, 5);
+}
+
+bool summ_bwd_tc_supported(const Dims& d, int dtype) {
+  return dtype == MUSE_BF16 && d.D == sb::D && d.Cq % 8 == 0;
+}
+
+int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
+
+int summ_bwd_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* off_q, const float* qbar,
+                const float* mu, const void* dkappa, const void* dnu, const float* dS, float* dK_perm, float* dV_perm,
+                int* status, cudaStream_t st) {
+  CUtensorMap tdka, tdnu, tK, tV;
+  const uint64_t grows = (uint64_t)d.B * d.Hq * d.SB * d.Cq, gcols = (uint64_t)d.Ck * sb::D;
+  int rc = make_tmap_bf16_pitched(&tdka, dkappa, grows, gcols, gcols * 2, sb::TI);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_pitched(&tdnu, dnu, grows, gcols, gcols * 2, sb::TI);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tK, Kp, (uint64_t)d.B * d.Hkv * d.N, sb::D, sb::NU);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tV, Vp, (uint64_t)d.B * d.Hkv * d.N, sb::D, sb::NU);
+  if (rc != MUSE_OK) return rc;
+  MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, sb::total));
+  prof_mark("k_summ_bwd_tc", st);
+  k_summ_bwd_tc<<<dim3(d.Ck, d.B * d.Hq), 128, sb::total, st>>>(d, tdka, tdnu, tK, tV, off_k, off_q, qbar, mu, dS, dK_perm,
+                                                                dV_perm, status);
+  MUSE_LAUNCH_OK();
+  return MUSE_OK;
+}
+
+}  // namespace muse

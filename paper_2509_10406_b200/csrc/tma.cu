@@ -35,4 +35,18 @@ int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t
   return r == CUDA_SUCCESS ? MUSE_OK : MUSE_ERR_CUDA;
 }
 
+// Same, for a matrix whose rows are `pitch_bytes` apart (a multiple of 16 bytes).
+int make_tmap_bf16_pitched(void* out_map, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr) return MUSE_ERR_CUDA;
+  cuuint64_t gdim[2] = {cols, rows};
+  cuuint64_t gstride[1] = {pitch_bytes};
+  cuuint32_t box[2] = {64, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(reinterpret_cast<CUtensorMap*>(out_map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base),
+                  gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MUSE_OK : MUSE_ERR_CUDA;
+}
+
 }  // namespace muse
