@@ -128,6 +128,9 @@ int bucket_sort(int, const int32_t* assign, int problems, int N, int C, int S, i
 // ---------------------------------------------------------------------------------------------
 // Lloyd iterations
 // ---------------------------------------------------------------------------------------------
+int assign_tc(const void* X, int problems, int N, int D, int C, const float* centres, const float* cnorm, void* chi,
+              void* clo, int32_t* assign, int* status, cudaStream_t st);
+
 __device__ __forceinline__ uint64_t splitmix64(uint64_t x) {
   uint64_t z = x + 0x9E3779B97F4A7C15ull;
   z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
@@ -317,10 +320,15 @@ static int lloyd_t(const Dims& d, const T* X, int problems, int C, int kind, con
                    int init_mode, uint64_t seed, int T_iters, int32_t* assign, float* centres, void* ws,
                    cudaStream_t st) {
   Arena ar(ws);
+  int32_t* status = ar.take<int32_t>(64);      // ws[0]: non-zero if a bounded device-side wait gave up
   float* cnorm = ar.take<float>((size_t)problems * C);
   int32_t* off = ar.take<int32_t>((size_t)problems * (C * d.S + 1));
   int32_t* perm = ar.take<int32_t>((size_t)problems * d.N);
   int32_t* scratch = ar.take<int32_t>((size_t)problems * sort_ws_elems(d.N, C * d.S));
+  __nv_bfloat16* chi = ar.take<__nv_bfloat16>((size_t)problems * C * D);
+  __nv_bfloat16* clo = ar.take<__nv_bfloat16>((size_t)problems * C * D);
+  constexpr bool kTensor = sizeof(T) == 2;     // bf16 inputs: distances on the tensor cores
+  MUSE_CUDA_OK(cudaMemsetAsync(status, 0, 64 * sizeof(int32_t), st));
   if (init_mode != MUSE_INIT_CENTRES) {
     prof_mark("k_init_centres", st);
     k_init_centres<T><<<dim3(C, problems), 32, 0, st>>>(X, d.N, D, C, init_idx, init_mode, seed, kind, centres);
@@ -333,9 +341,14 @@ static int lloyd_t(const Dims& d, const T* X, int problems, int C, int kind, con
   const size_t smem = (size_t)((kAsgRows + kAsgCols) * (D + 4) + kAsgCols) * sizeof(float);
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_assign<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   for (int it = 0; it <= T_iters; ++it) {
-    prof_mark("k_assign", st);
-    k_assign<T, D><<<dim3(cdiv(d.N, kAsgRows), problems), kAsgThreads, smem, st>>>(X, d.N, C, centres, cnorm, assign);
-    MUSE_LAUNCH_OK();
+    if (kTensor) {
+      int rc = assign_tc(X, problems, d.N, D, C, centres, cnorm, chi, clo, assign, status, st);
+      if (rc != MUSE_OK) return rc;
+    } else {
+      prof_mark("k_assign", st);
+      k_assign<T, D><<<dim3(cdiv(d.N, kAsgRows), problems), kAsgThreads, smem, st>>>(X, d.N, C, centres, cnorm, assign);
+      MUSE_LAUNCH_OK();
+    }
     if (it == T_iters) break;
     int rc = bucket_sort(0, assign, problems, d.N, C, d.S, d.Bs, kind, off, perm, scratch, st);
     if (rc != MUSE_OK) return rc;
@@ -348,10 +361,13 @@ static int lloyd_t(const Dims& d, const T* X, int problems, int C, int kind, con
 
 size_t lloyd_ws_bytes(const Dims& d, int problems, int C, int) {
   Arena ar(nullptr);
+  ar.take<int32_t>(64);
   ar.take<float>((size_t)problems * C);
   ar.take<int32_t>((size_t)problems * (C * d.S + 1));
   ar.take<int32_t>((size_t)problems * d.N);
   ar.take<int32_t>((size_t)problems * sort_ws_elems(d.N, C * d.S));
+  ar.take<__nv_bfloat16>((size_t)problems * C * d.D);
+  ar.take<__nv_bfloat16>((size_t)problems * C * d.D);
   return ar.used;
 }
 
