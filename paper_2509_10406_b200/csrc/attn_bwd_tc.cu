@@ -191,6 +191,8 @@ k_local_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
   bwd_teardown(c, RowsSmem<D>::cols, tid, status);
 }
 
+constexpr int kRetSplitRows = 4;      // CTAs sharing the 128-pair tiles of one (cluster, plane) group
+
 template <int D>
 __global__ void __launch_bounds__(128)
 k_ret_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO, const bf16* __restrict__ Kp,
@@ -202,12 +204,12 @@ k_ret_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO
   __shared__ uint32_t tbase_s;
   __shared__ int32_t pid_s[kBM];
   const int tid = threadIdx.x;
-  const int j = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z;
+  const int j = blockIdx.x, pl = blockIdx.y / kRetSplitRows, sub = blockIdx.y % kRetSplitRows, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
   const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)pl * dm.Ck + j;
   const int g0 = go[0], g1 = go[1];
-  if (g0 >= g1) return;
+  if (g0 + sub * kBM >= g1) return;                   // this split has no pair tile
   const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const int k0 = ok[0], k1 = ok[pl + 1];
   BwdCtx c;
@@ -215,7 +217,7 @@ k_ret_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO
   const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
   const bf16* Kb = Kp + (size_t)pk * dm.N * D; const bf16* Vb = Vp + (size_t)pk * dm.N * D;
   const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
-  for (int t0 = g0; t0 < g1 && c.ok; t0 += kBM) {
+  for (int t0 = g0 + sub * kBM; t0 < g1 && c.ok; t0 += kRetSplitRows * kBM) {
     const int nq = min(kBM, g1 - t0);
     __syncthreads();
     pid_s[tid] = tid < nq ? pr[t0 + tid] : 0;
@@ -348,8 +350,27 @@ k_local_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict_
   bwd_teardown(c, SM::cols, tid, status);
 }
 
-// One CTA per (key cluster j, head): 128-key tiles of the cluster's visible run; every plane that
-// sees a tile feeds its retrieving pairs 64 at a time.
+// One CTA per (key cluster j, plane, split, head): 128-key tiles of the run the plane sees, fed with
+// every kRetSplit-th tile of 64 retrieving pairs.  Popular clusters are retrieved by thousands of
+// queries, so the pair tiles are spread over kRetSplit CTAs and over the planes; each CTA adds
+// its partial dK, dV with vector float atomics into the zero-initialised accumulators.
+constexpr int kRetSplit = 8;
+
+template <int D>
+__device__ __forceinline__ void add_acc_row(const BwdCtx& c, uint32_t col, float f, float* __restrict__ dst, bool write, int tid) {
+  const uint32_t t = c.tbase + ((uint32_t)((tid >> 5) * 32) << 16) + col;
+#pragma unroll
+  for (int d0 = 0; d0 < D; d0 += 32) {
+    float v[32];
+    tc::tmem_ld32(t + d0, v);
+    if (write) {
+#pragma unroll
+      for (int i = 0; i < 32; i += 4)
+        atomicAdd(reinterpret_cast<float4*>(dst + d0 + i), make_float4(v[i] * f, v[i + 1] * f, v[i + 2] * f, v[i + 3] * f));
+    }
+  }
+}
+
 template <int D>
 __global__ void __launch_bounds__(128)
 k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO, const bf16* __restrict__ Kp,
@@ -363,15 +384,14 @@ k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
   __shared__ float Ls[kBN], ds[kBN];
   __shared__ int32_t tok_s[kBN];
   const int tid = threadIdx.x;
-  const int j = blockIdx.x, pq = blockIdx.y;
+  const int j = blockIdx.x, pl = blockIdx.y / kRetSplit, sub = blockIdx.y % kRetSplit, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
-  const int32_t* go = goff + (size_t)pq * (nkeys + 1);
+  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)pl * dm.Ck + j;
   const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
-  const int kbeg = ok[0], kvis = ok[dm.SB];
-  int total_pairs = 0;
-  for (int pl = 0; pl < dm.SB; ++pl) total_pairs += go[(size_t)pl * dm.Ck + j + 1] - go[(size_t)pl * dm.Ck + j];
-  if (kbeg >= kvis || total_pairs == 0) return;
+  const int kbeg = ok[0], kvis = ok[pl + 1];
+  const int g0 = go[0], g1 = go[1], ntiles = (g1 - g0 + kBN - 1) / kBN;
+  if (kbeg >= kvis || sub >= ntiles) return;          // nothing for this (plane, split): no TMEM taken
   BwdCtx c;
   bwd_setup(c, sm_raw, bar, &tbase_s, SM::cols, tid);
   const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
@@ -383,30 +403,25 @@ k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
     fill_tile<D, kBM>(c.sm + SM::k, nkc, [&](int r) { return Kb + (size_t)(c0 + r) * D; }, tid);
     fill_tile<D, kBM>(c.sm + SM::v, nkc, [&](int r) { return Vb + (size_t)(c0 + r) * D; }, tid);
     bool started = false;
-    for (int pl = 0; pl < dm.SB && c.ok; ++pl) {
-      const int vis_end = ok[pl + 1];
-      if (c0 >= vis_end) continue;
-      const bool mine = c0 + tid < vis_end;                // this thread's key is visible to the plane
-      const int g0 = go[(size_t)pl * dm.Ck + j], g1 = go[(size_t)pl * dm.Ck + j + 1];
-      for (int t0 = g0; t0 < g1 && c.ok; t0 += kBN) {
-        const int nq = min(kBN, g1 - t0);
-        __syncthreads();
-        if (tid < kBN) {
-          const int tok = tid < nq ? pr[t0 + tid] / dm.m : 0;
-          tok_s[tid] = tok;
-          Ls[tid] = tid < nq ? LSE[(size_t)pq * dm.N + tok] * kLog2e : 0.f;
-          ds[tid] = tid < nq ? delta[(size_t)pq * dm.N + tok] : 0.f;
-        }
-        __syncthreads();
-        fill_tile<D, kBN>(c.sm + SM::q, nq, [&](int r) { return Qb + (size_t)tok_s[r] * D; }, tid);
-        fill_tile<D, kBN>(c.sm + SM::dO, nq, [&](int r) { return dOb + (size_t)tok_s[r] * D; }, tid);
-        dkdv_step_tc<D>(c, Ls, ds, [&](int col) { return col < nq && mine; }, dm.sigma * kLog2e, started, tid);
+    const bool mine = tid < nkc;
+    for (int t = sub; t < ntiles && c.ok; t += kRetSplit) {
+      const int t0 = g0 + t * kBN, nq = min(kBN, g1 - t0);
+      __syncthreads();
+      if (tid < kBN) {
+        const int tok = tid < nq ? pr[t0 + tid] / dm.m : 0;
+        tok_s[tid] = tok;
+        Ls[tid] = tid < nq ? LSE[(size_t)pq * dm.N + tok] * kLog2e : 0.f;
+        ds[tid] = tid < nq ? delta[(size_t)pq * dm.N + tok] : 0.f;
       }
+      __syncthreads();
+      fill_tile<D, kBN>(c.sm + SM::q, nq, [&](int r) { return Qb + (size_t)tok_s[r] * D; }, tid);
+      fill_tile<D, kBN>(c.sm + SM::dO, nq, [&](int r) { return dOb + (size_t)tok_s[r] * D; }, tid);
+      dkdv_step_tc<D>(c, Ls, ds, [&](int col) { return col < nq && mine; }, dm.sigma * kLog2e, started, tid);
     }
     if (c.ok && started) {
       const size_t row = ((size_t)pq * dm.N + c0 + tid) * D;
-      read_acc_row<D>(c, 2 * kBN, 1.f, dV_perm + row, tid < nkc, tid);
-      read_acc_row<D>(c, 2 * kBN + D, dm.sigma, dK_perm + row, tid < nkc, tid);
+      add_acc_row<D>(c, 2 * kBN, 1.f, dV_perm + row, tid < nkc, tid);
+      add_acc_row<D>(c, 2 * kBN + D, dm.sigma, dK_perm + row, tid < nkc, tid);
     }
     tc::fence_before_sync();
   }
@@ -444,10 +459,10 @@ int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, con
                float* dK_perm, float* dV_perm, int* status, cudaStream_t st) {
   const int pq = d.B * d.Hq;
   prof_mark("k_ret_bwd_dkdv_tc", st);
-  MUSE_TC_LAUNCH(k_ret_bwd_dkdv_tc, KeysSmem, dim3(d.Ck, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
+  MUSE_TC_LAUNCH(k_ret_bwd_dkdv_tc, KeysSmem, dim3(d.Ck, d.SB * kRetSplit, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
                  (const bf16*)Vp, LSE, delta, off_k, goff, pairs, dK_perm, dV_perm, status);
   prof_mark("k_ret_bwd_dq_tc", st);
-  MUSE_TC_LAUNCH(k_ret_bwd_dq_tc, RowsSmem, dim3(d.Ck, d.SB, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
+  MUSE_TC_LAUNCH(k_ret_bwd_dq_tc, RowsSmem, dim3(d.Ck, d.SB * kRetSplitRows, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
                  (const bf16*)Vp, LSE, delta, off_k, goff, pairs, dq_part, status);
   return MUSE_OK;
 }

@@ -201,6 +201,10 @@ k_local_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ K, 
 }
 
 // ---- exact retrieval ---------------------------------------------------------------------------------
+// A popular cluster is retrieved by thousands of queries of a block: its 128-pair tiles are
+// spread over kRetFwdSplit CTAs.
+constexpr int kRetFwdSplit = 4;
+
 template <int D>
 __global__ void __launch_bounds__(128)
 k_ret_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, const bf16* __restrict__ Vp,
@@ -211,12 +215,12 @@ k_ret_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, c
   __shared__ uint32_t tbase_s;
   __shared__ int32_t pid_s[kTcM];
   const int tid = threadIdx.x;
-  const int j = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z;
+  const int j = blockIdx.x, pl = blockIdx.y / kRetFwdSplit, sub = blockIdx.y % kRetFwdSplit, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
   const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)pl * dm.Ck + j;
   const int g0 = go[0], g1 = go[1];
-  if (g0 >= g1) return;                                  // before any TMEM allocation
+  if (g0 + sub * kTcM >= g1) return;                     // no pair tile for this split (before any TMEM allocation)
   const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const int k0 = ok[0], k1 = ok[pl + 1];
   TcCtx c;
@@ -226,7 +230,7 @@ k_ret_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, c
   const bf16* Vb = Vp + (size_t)pk * dm.N * D;
   const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
   const float scale2 = dm.sigma * 1.4426950408889634f;
-  for (int t0 = g0; t0 < g1 && c.ok; t0 += kTcM) {
+  for (int t0 = g0 + sub * kTcM; t0 < g1 && c.ok; t0 += kRetFwdSplit * kTcM) {
     const int nq = min(kTcM, g1 - t0);
     __syncthreads();
     pid_s[tid] = tid < nq ? pr[t0 + tid] : 0;
@@ -266,7 +270,7 @@ int local_fwd_tc(const Dims& d, const void* Q, const void* K, const void* V, flo
 
 int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
                const int32_t* pairs, float* o_part, float* l_part, int* status, cudaStream_t st) {
-  dim3 grid(d.Ck, d.SB, d.B * d.Hq);
+  dim3 grid(d.Ck, d.SB * kRetFwdSplit, d.B * d.Hq);
   prof_mark("k_ret_fwd_tc", st);
   if (d.D == 128) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdTcSmem<128>::total));
