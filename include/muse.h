@@ -113,6 +113,27 @@ MUSE_API int muse_cluster(const muse_params_t* p, const void* Q, const void* K,
                  int32_t* assign_q, int32_t* assign_k, float* qbar, float* kcent,
                  void* ws, size_t ws_bytes, cudaStream_t stream);
 
+/* Clustering without a caller-provided workspace (the paper has no counterpart; this is a
+ * deployment aid).  Same inputs, outputs and results as muse_cluster, but the scratch memory is
+ * a fixed 32 MiB array built into the library's device image, so the call performs no device
+ * allocation of any kind and needs no scratch pointer.  It is meant for callers that cannot
+ * allocate or own no spare device memory: code running inside a serving loop where a device
+ * allocation would stall every stream, plugins living under a framework whose pool already
+ * owns the whole GPU, or hosts that must not fail with out-of-memory in mid-request.
+ *   - Every GPU that loads the library carries the 32 MiB until the process exits.
+ *   - Problems whose clustering scratch (muse_workspace_bytes out[0]) exceeds
+ *     muse_cluster_noalloc_max_bytes() are rejected with MUSE_ERR_WORKSPACE; nothing is launched.
+ *   - The first call on each device looks up the array's device address (the device must be
+ *     current); make that first call outside any stream capture.
+ *   - All calls share the one array and find in it whatever the previous call left; the stage
+ *     clears what it needs zeroed itself.  Two calls that overlap on the GPU (different streams,
+ *     or different threads) race on it: serialise them. */
+MUSE_API int muse_cluster_noalloc(const muse_params_t* p, const void* Q, const void* K,
+                         const int32_t* init_q, const int32_t* init_k,
+                         int32_t* assign_q, int32_t* assign_k, float* qbar, float* kcent,
+                         cudaStream_t stream);
+MUSE_API size_t muse_cluster_noalloc_max_bytes(void);
+
 /* Buckets the keys by (cluster, block) and builds the accumulated tilted summaries
  * mu_ijb = log sum exp(sigma qbar_i.k), kappa_ijb, nu_ijb = weighted means of k, v over the
  * keys of cluster j in blocks < b (Eq. 3-5 and "Causal accumulation").

@@ -21,7 +21,8 @@ MUSE_SEL_PER_QUERY, MUSE_SEL_PER_QCLUSTER = 0, 1
 MUSE_INIT_INDICES, MUSE_INIT_STRIDED, MUSE_INIT_CENTRES = 0, 1, 2
 
 EXPORTS = ("muse_workspace_bytes", "muse_summaries_layout", "muse_cluster", "muse_summarize",
-           "muse_attn_fwd", "muse_attn_bwd", "muse_profile", "muse_profile_report", "muse_strerror")
+           "muse_attn_fwd", "muse_attn_bwd", "muse_cluster_noalloc", "muse_cluster_noalloc_max_bytes",
+           "muse_profile", "muse_profile_report", "muse_strerror")
 
 
 class MuseParams(ctypes.Structure):
@@ -83,11 +84,14 @@ def lib() -> ctypes.CDLL:
         L.muse_attn_fwd.argtypes = [pp, vp, vp, vp, i32p, f32p, i32p, i32p, vp, i32p, vp, f32p, i32p, vp, sz, vp]
         L.muse_attn_bwd.argtypes = [pp, vp, vp, vp, vp, f32p, vp, i32p, f32p, i32p, i32p, vp, i32p, vp, vp, vp,
                                     vp, sz, vp]
+        L.muse_cluster_noalloc.argtypes = [pp, vp, vp, i32p, i32p, i32p, i32p, f32p, f32p, vp]
+        L.muse_cluster_noalloc_max_bytes.argtypes = []
         L.muse_profile.argtypes = [ctypes.c_int]
         L.muse_profile_report.argtypes = [ctypes.c_char_p, sz]
         for name in EXPORTS[:-1]:
             getattr(L, name).restype = ctypes.c_int
         L.muse_profile_report.restype = ctypes.c_long
+        L.muse_cluster_noalloc_max_bytes.restype = ctypes.c_size_t
         _lib = L
     return _lib
 
@@ -147,6 +151,19 @@ def muse_cluster(p, Q, K, init_q, init_k, assign_q, assign_k, qbar, kcent, ws):
     _check(lib().muse_cluster(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(init_q), _ptr(init_k), _ptr(assign_q),
                               _ptr(assign_k), _ptr(qbar), _ptr(kcent), _ptr(ws), ws.numel() * ws.element_size(),
                               _stream()), "muse_cluster")
+
+
+def muse_cluster_noalloc(p, Q, K, init_q, init_k, assign_q, assign_k, qbar, kcent):
+    """muse_cluster on the library's built-in 32 MiB scratch: no workspace argument, no device
+    allocation.  For callers that may not allocate (see include/muse.h); raises MuseError with
+    'workspace too small' when the problem needs more scratch than the built-in array holds.
+    Calls that overlap on the GPU share the array and must be serialised by the caller."""
+    _check(lib().muse_cluster_noalloc(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(init_q), _ptr(init_k), _ptr(assign_q),
+                                      _ptr(assign_k), _ptr(qbar), _ptr(kcent), _stream()), "muse_cluster_noalloc")
+
+
+def muse_cluster_noalloc_max_bytes() -> int:
+    return int(lib().muse_cluster_noalloc_max_bytes())
 
 
 def muse_summarize(p, K, V, assign_k, qbar, off_k, perm_k, summaries, ws):
