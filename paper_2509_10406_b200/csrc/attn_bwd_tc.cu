@@ -28,6 +28,28 @@ __device__ __forceinline__ void fill_tile(unsigned char* dst, int n, RowPtr row_
   }
 }
 
+// A [ROWS][D] tile held in registers between its global loads and its shared-memory stores, so
+// that the loads of the next tile are in flight while the tensor core works on the current one.
+template <int D, int ROWS> struct TileRegs { static constexpr int N = ROWS * (D / 8) / 128; uint4 v[N]; };
+template <int D, int ROWS, class RowPtr>
+__device__ __forceinline__ void tile_ldg(TileRegs<D, ROWS>& t, int n, RowPtr row_ptr, int tid) {
+  constexpr int CPR = D / 8;
+#pragma unroll
+  for (int k = 0; k < TileRegs<D, ROWS>::N; ++k) {
+    const int e = tid + 128 * k, r = e / CPR, ck = e % CPR;
+    t.v[k] = r < n ? __ldg(reinterpret_cast<const uint4*>(row_ptr(r)) + ck) : make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+template <int D, int ROWS>
+__device__ __forceinline__ void tile_sts(const TileRegs<D, ROWS>& t, unsigned char* dst, int tid) {
+  constexpr int CPR = D / 8;
+#pragma unroll
+  for (int k = 0; k < TileRegs<D, ROWS>::N; ++k) {
+    const int e = tid + 128 * k, r = e / CPR, ck = e % CPR;
+    *reinterpret_cast<uint4*>(dst + (ck >> 3) * ROWS * 128 + tc::sw128_off(r, ck & 7)) = t.v[k];
+  }
+}
+
 // K-major view of a [ROWS][D] tile at k-step ks (16 elements of D)
 template <int ROWS> __device__ __forceinline__ uint64_t desc_k(uint32_t base, int ks) {
   return tc::smem_desc_sw128(base + (ks / 4) * ROWS * 128 + (ks % 4) * 32, 16, 1024);
@@ -94,10 +116,15 @@ __device__ __forceinline__ bool dq_rows_tc(BwdCtx& c, const bf16* __restrict__ K
                  va = tc::smem_u32(c.sm + SM::v), ga = tc::smem_u32(c.sm + SM::g);
   const int my_limit = limit(tid);
   bool first = true;
+  TileRegs<D, kBN> kreg, vreg;
+  if (k_lo < k_hi) {
+    tile_ldg<D, kBN>(kreg, min(kBN, k_hi - k_lo), [&](int r) { return Kb + (size_t)(k_lo + r) * D; }, tid);
+    tile_ldg<D, kBN>(vreg, min(kBN, k_hi - k_lo), [&](int r) { return Vb + (size_t)(k_lo + r) * D; }, tid);
+  }
   for (int c0 = k_lo; c0 < k_hi && c.ok; c0 += kBN) {
     const int nk = min(kBN, k_hi - c0);
-    fill_tile<D, kBN>(c.sm + SM::k, nk, [&](int r) { return Kb + (size_t)(c0 + r) * D; }, tid);
-    fill_tile<D, kBN>(c.sm + SM::v, nk, [&](int r) { return Vb + (size_t)(c0 + r) * D; }, tid);
+    tile_sts<D, kBN>(kreg, c.sm + SM::k, tid);
+    tile_sts<D, kBN>(vreg, c.sm + SM::v, tid);
     tc::fence_async_smem();
     tc::fence_before_sync();
     __syncthreads();
@@ -109,6 +136,11 @@ __device__ __forceinline__ bool dq_rows_tc(BwdCtx& c, const bf16* __restrict__ K
 #pragma unroll
       for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase + kBN, desc_k<kBM>(da, ks), desc_k<kBN>(va, ks), idesc, ks > 0);
       tc::mma_commit(&c.bar[0]);
+    }
+    if (c0 + kBN < k_hi) {                   // next key tile: loads fly while the MMAs and the softmax piece run
+      const int cn = c0 + kBN, nn = min(kBN, k_hi - cn);
+      tile_ldg<D, kBN>(kreg, nn, [&](int r) { return Kb + (size_t)(cn + r) * D; }, tid);
+      tile_ldg<D, kBN>(vreg, nn, [&](int r) { return Vb + (size_t)(cn + r) * D; }, tid);
     }
     if (!tc::mbar_wait(&c.bar[0], c.ph0)) { c.ok = false; break; }
     c.ph0 ^= 1;
@@ -249,9 +281,9 @@ template <int D> struct KeysSmem {
 // One tile of 64 query rows (already in shared memory with their L2 / delta in Ls / ds).
 // valid(u_row) = number of leading query columns ... see callers: mask(col) tells whether
 // query column `col` sees this thread's key.
-template <int D, class Mask>
+template <int D, class Mask, class Prefetch>
 __device__ __forceinline__ void dkdv_step_tc(BwdCtx& c, const float* __restrict__ Ls, const float* __restrict__ ds,
-                                             Mask mask, float scale2, bool& started, int tid) {
+                                             Mask mask, float scale2, bool& started, int tid, Prefetch prefetch) {
   typedef KeysSmem<D> SM;
   const int warp = tid >> 5;
   const uint32_t t_s = c.tbase + ((uint32_t)(warp * 32) << 16), t_dp = t_s + kBN;
@@ -269,6 +301,7 @@ __device__ __forceinline__ void dkdv_step_tc(BwdCtx& c, const float* __restrict_
     for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase + kBN, desc_k<kBM>(va, ks), desc_k<kBN>(da, ks), idesc, ks > 0);
     tc::mma_commit(&c.bar[0]);
   }
+  prefetch();                                  // global loads of the next query tile, overlapped with the MMAs
   if (!tc::mbar_wait(&c.bar[0], c.ph0)) { c.ok = false; return; }
   c.ph0 ^= 1;
   tc::fence_after_sync();
@@ -332,15 +365,25 @@ k_local_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict_
   fill_tile<D, kBM>(c.sm + SM::v, nk, [&](int r) { return Vb + (size_t)(k0 + r) * D; }, tid);
   bool started = false;
   const int u = k0 + tid;
+  TileRegs<D, kBN> qreg, oreg;
+  float Lreg = 0.f, dreg = 0.f;
+  auto load_q = [&](int q0) {
+    const int nq = min(kBN, bend - q0);
+    tile_ldg<D, kBN>(qreg, nq, [&](int r) { return Qb + (size_t)(q0 + r) * D; }, tid);
+    tile_ldg<D, kBN>(oreg, nq, [&](int r) { return dOb + (size_t)(q0 + r) * D; }, tid);
+    if (tid < kBN) {
+      Lreg = tid < nq ? LSE[(size_t)pq * dm.N + q0 + tid] * kLog2e : 0.f;
+      dreg = tid < nq ? delta[(size_t)pq * dm.N + q0 + tid] : 0.f;
+    }
+  };
+  load_q(k0);
   for (int q0 = k0; q0 < bend && c.ok; q0 += kBN) {
     const int nq = min(kBN, bend - q0);
-    fill_tile<D, kBN>(c.sm + SM::q, nq, [&](int r) { return Qb + (size_t)(q0 + r) * D; }, tid);
-    fill_tile<D, kBN>(c.sm + SM::dO, nq, [&](int r) { return dOb + (size_t)(q0 + r) * D; }, tid);
-    if (tid < kBN) {
-      Ls[tid] = tid < nq ? LSE[(size_t)pq * dm.N + q0 + tid] * kLog2e : 0.f;
-      ds[tid] = tid < nq ? delta[(size_t)pq * dm.N + q0 + tid] : 0.f;
-    }
-    dkdv_step_tc<D>(c, Ls, ds, [&](int col) { return col < nq && tid < nk && u <= q0 + col; }, dm.sigma * kLog2e, started, tid);
+    tile_sts<D, kBN>(qreg, c.sm + SM::q, tid);
+    tile_sts<D, kBN>(oreg, c.sm + SM::dO, tid);
+    if (tid < kBN) { Ls[tid] = Lreg; ds[tid] = dreg; }
+    dkdv_step_tc<D>(c, Ls, ds, [&](int col) { return col < nq && tid < nk && u <= q0 + col; }, dm.sigma * kLog2e, started, tid,
+                    [&]() { if (q0 + kBN < bend) load_q(q0 + kBN); });
   }
   if (c.ok) {
     const size_t row = ((size_t)pq * dm.N + k0 + tid) * D;
@@ -404,19 +447,26 @@ k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
     fill_tile<D, kBM>(c.sm + SM::v, nkc, [&](int r) { return Vb + (size_t)(c0 + r) * D; }, tid);
     bool started = false;
     const bool mine = tid < nkc;
+    TileRegs<D, kBN> qreg, oreg;
+    float Lreg = 0.f, dreg = 0.f;
+    auto load_pairs = [&](int t) {             // gathers the rows of pair tile t (token = pair id / m)
+      const int t0 = g0 + t * kBN, nq = min(kBN, g1 - t0);
+      tile_ldg<D, kBN>(qreg, nq, [&](int r) { return Qb + (size_t)(__ldg(pr + t0 + r) / dm.m) * D; }, tid);
+      tile_ldg<D, kBN>(oreg, nq, [&](int r) { return dOb + (size_t)(__ldg(pr + t0 + r) / dm.m) * D; }, tid);
+      if (tid < kBN) {
+        const int tok = tid < nq ? __ldg(pr + t0 + tid) / dm.m : 0;
+        Lreg = tid < nq ? LSE[(size_t)pq * dm.N + tok] * kLog2e : 0.f;
+        dreg = tid < nq ? delta[(size_t)pq * dm.N + tok] : 0.f;
+      }
+    };
+    load_pairs(sub);
     for (int t = sub; t < ntiles && c.ok; t += kRetSplit) {
       const int t0 = g0 + t * kBN, nq = min(kBN, g1 - t0);
-      __syncthreads();
-      if (tid < kBN) {
-        const int tok = tid < nq ? pr[t0 + tid] / dm.m : 0;
-        tok_s[tid] = tok;
-        Ls[tid] = tid < nq ? LSE[(size_t)pq * dm.N + tok] * kLog2e : 0.f;
-        ds[tid] = tid < nq ? delta[(size_t)pq * dm.N + tok] : 0.f;
-      }
-      __syncthreads();
-      fill_tile<D, kBN>(c.sm + SM::q, nq, [&](int r) { return Qb + (size_t)tok_s[r] * D; }, tid);
-      fill_tile<D, kBN>(c.sm + SM::dO, nq, [&](int r) { return dOb + (size_t)tok_s[r] * D; }, tid);
-      dkdv_step_tc<D>(c, Ls, ds, [&](int col) { return col < nq && mine; }, dm.sigma * kLog2e, started, tid);
+      tile_sts<D, kBN>(qreg, c.sm + SM::q, tid);
+      tile_sts<D, kBN>(oreg, c.sm + SM::dO, tid);
+      if (tid < kBN) { Ls[tid] = Lreg; ds[tid] = dreg; }
+      dkdv_step_tc<D>(c, Ls, ds, [&](int col) { return col < nq && mine; }, dm.sigma * kLog2e, started, tid,
+                      [&]() { if (t + kRetSplit < ntiles) load_pairs(t + kRetSplit); });
     }
     if (c.ok && started) {
       const size_t row = ((size_t)pq * dm.N + c0 + tid) * D;
