@@ -641,7 +641,7 @@ int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, con
 bool far_bwd_tc_supported(const Dims& d, int dtype);
 int far_bwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const void* dO, const float* qbar, const float* LSE,
                const float* delta, const int32_t* off_q, const int32_t* perm_q, const int32_t* sel, float* dQacc,
-               void* dkappa, void* dnu, float* dS, int* status, cudaStream_t st);
+               void* dkappa, void* dnu, float* dS, int grad_by_key_cluster, int* status, cudaStream_t st);
 
 bool summ_bwd_tc_supported(const Dims& d, int dtype);
 int summ_bwd_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* off_q, const float* qbar,
@@ -739,8 +739,9 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
     }
     const bool far_tc = far_bwd_tc_supported(d, dtype) && getenv("MUSE_FAR_SIMT") == nullptr;
     const size_t fsm = (size_t)(4 * kTile * (D + 4) + kTile * kLDP) * sizeof(float) + (size_t)kTile * cdiv(d.Ck, 32) * sizeof(uint32_t);
+    const bool summ_tc = far_tc && summ_bwd_tc_supported(d, dtype) && getenv("MUSE_SUMM_SIMT") == nullptr;
     if (far_tc) {
-      rc = far_bwd_tc(d, sp, Q, dO, qbar, LSE, w.delta, w.off_q, w.perm_q, sel, w.dQacc, w.dkappa, w.dnu, w.dS, w.status, st);
+      rc = far_bwd_tc(d, sp, Q, dO, qbar, LSE, w.delta, w.off_q, w.perm_q, sel, w.dQacc, w.dkappa, w.dnu, w.dS, summ_tc ? 1 : 0, w.status, st);
       if (rc != MUSE_OK) return rc;
     } else {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fsm));
@@ -750,7 +751,7 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
     MUSE_LAUNCH_OK();
     }
     const size_t ssm = (size_t)(5 * kTile * (D + 4) + kTile * kLDP) * sizeof(float);
-    if (far_tc && summ_bwd_tc_supported(d, dtype) && getenv("MUSE_SUMM_SIMT") == nullptr) {
+    if (summ_tc) {
       rc = summ_bwd_tc(d, Kp, Vp, off_k, w.off_q, qbar, mu, w.dkappa, w.dnu, w.dS, w.dK_perm, w.dV_perm, w.status, st);
       if (rc != MUSE_OK) return rc;
     } else if (far_tc) {

@@ -34,7 +34,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
              const float* __restrict__ qbar, const float* __restrict__ LSE, const float* __restrict__ delta,
              const int32_t* __restrict__ off_q, const int32_t* __restrict__ perm_q, const int32_t* __restrict__ sel,
              const float* __restrict__ beta, float* __restrict__ dQacc, bf16* __restrict__ dkappa,
-             bf16* __restrict__ dnu, float* __restrict__ dS, int* __restrict__ status) {
+             bf16* __restrict__ dnu, float* __restrict__ dS, int grad_by_key_cluster, int* __restrict__ status) {
   using namespace fb;
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar_full, bar1, bar2;
@@ -192,7 +192,10 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       __syncthreads();
       const float gtot = part[0][L] + part[1][L];
       float dot = 0.f;
-      bf16* dst = (wg == 0 ? dnu : dkappa) + (ent0 + j) * D;
+      // gradient entry: [plane][i][j] like the summaries, or [plane][j][i] so that the key-side
+      // pass finds the 128 query clusters of one key cluster in one contiguous tile
+      const size_t gent = grad_by_key_cluster ? (((size_t)pq * dm.SB + pl) * Ck + j) * dm.Cq + i : ent0 + j;
+      bf16* dst = (wg == 0 ? dnu : dkappa) + gent * D;
 #pragma unroll
       for (int d0 = 0; d0 < D; d0 += 32) {
         float v[32];
@@ -226,7 +229,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       tc::fence_async_smem();          // generic reads of the tiles are ordered before the next TMA writes
       tc::fence_before_sync();
       __syncthreads();
-      if (wg == 0 && ok) dS[ent0 + j] = gtot - dots[0][L] - dots[1][L];
+      if (wg == 0 && ok) dS[gent] = gtot - dots[0][L] - dots[1][L];
     }
     // ---- dq: warpgroup p reads pass p (thread = output dim), adds into the fp32 accumulator
     for (int p = wg; p < np; p += 2) {
@@ -257,7 +260,7 @@ bool far_bwd_tc_supported(const Dims& d, int dtype) {
 
 int far_bwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const void* dO, const float* qbar, const float* LSE,
                const float* delta, const int32_t* off_q, const int32_t* perm_q, const int32_t* sel, float* dQacc,
-               void* dkappa, void* dnu, float* dS, int* status, cudaStream_t st) {
+               void* dkappa, void* dnu, float* dS, int grad_by_key_cluster, int* status, cudaStream_t st) {
   const uint64_t ent = (uint64_t)d.B * d.Hq * d.SB * d.Cq * d.Ck;
   CUtensorMap khi, klo, nu;
   int rc = make_tmap_bf16_rows(&khi, sp.khi, ent, fb::D, fb::TJ);
@@ -269,7 +272,7 @@ int far_bwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const void* dO,
   prof_mark("k_far_bwd_tc", st);
   k_far_bwd_tc<<<dim3(d.Cq, d.SB, d.B * d.Hq), fb::THREADS, smem, st>>>(
       d, khi, klo, nu, (const bf16*)Q, (const bf16*)dO, qbar, LSE, delta, off_q, perm_q, sel, sp.beta, dQacc, (bf16*)dkappa,
-      (bf16*)dnu, dS, status);
+      (bf16*)dnu, dS, grad_by_key_cluster, status);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }

@@ -8,7 +8,9 @@
 // (the shared-memory qbar tiles already carry the factor sigma)
 // Query clusters sit on the MMA M side for the three D-contractions (one thread per i computes
 // w and w*c) and on the K side for the three i-contractions, whose outputs are transposed
-// ([d][u]) so that the read-out is coalesced over d.  Planes are handled independently.
+// ([d][u]) so that the read-out is coalesced over d.  Planes are handled independently and
+// accumulate, together with the query-cluster tiles, in tensor memory; the far-field backward
+// stores its gradients [plane][j][i] so that each (plane, j, 128 i) tile is one contiguous TMA box.
 #include <cuda.h>
 #include "common.cuh"
 #include "tc05.cuh"
@@ -60,62 +62,73 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
                  aDnu = tc::smem_u32(sm + oDnu), aK = tc::smem_u32(sm + oK), aV = tc::smem_u32(sm + oV),
                  aW = tc::smem_u32(sm + oW), aWc = tc::smem_u32(sm + oWc);
 
-  for (int i0 = 0; i0 < dm.Cq && ok; i0 += TI) {
-    // sigma * qbar tile as bf16 hi + lo (thread = row)
+  const int kvis = ok_[dm.SB];
+  for (int c0 = kbeg; c0 < kvis && ok; c0 += NU) {        // 64 keys of the cluster at a time (usually one chunk)
     __syncthreads();
-    {
-      const int i = i0 + tid;
-      const float* src = qbar + ((size_t)pq * dm.Cq + (i < dm.Cq ? i : 0)) * D;
-#pragma unroll
-      for (int ck = 0; ck < D / 8; ++ck) {
-        uint32_t wh[4], wl[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          float x0 = i < dm.Cq ? src[ck * 8 + 2 * e] * dm.sigma : 0.f, x1 = i < dm.Cq ? src[ck * 8 + 2 * e + 1] * dm.sigma : 0.f;
-          __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
-          __nv_bfloat162 ll = __floats2bfloat162_rn(x0 - __low2float(hh), x1 - __high2float(hh));
-          wh[e] = *reinterpret_cast<uint32_t*>(&hh); wl[e] = *reinterpret_cast<uint32_t*>(&ll);
-        }
-        const uint32_t off = (ck >> 3) * TI * 128 + tc::sw128_off(tid, ck & 7);
-        *reinterpret_cast<uint4*>(sm + oQhi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
-        *reinterpret_cast<uint4*>(sm + oQlo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
-      }
+    if (tid == 0) {
+      tc::mbar_expect_tx(&bar_kv, 2 * kKeys);
+      const int row = (int)((size_t)pk * dm.N + c0);
+      tc::tma_load_2d(sm + oK, &tm_K, 0, row, &bar_kv); tc::tma_load_2d(sm + oK + NU * 128, &tm_K, 64, row, &bar_kv);
+      tc::tma_load_2d(sm + oV, &tm_V, 0, row, &bar_kv); tc::tma_load_2d(sm + oV + NU * 128, &tm_V, 64, row, &bar_kv);
     }
-    for (int pl = 0; pl < dm.SB && ok; ++pl) {
-      const int kend = ok_[pl + 1];
-      if (kend <= kbeg) continue;                       // empty prefix: nothing was summarised
-      const int i = i0 + tid, blk = dm.causal ? pl + 1 : 0;
-      const size_t ent = (((size_t)pq * dm.SB + pl) * dm.Cq + (i < dm.Cq ? i : 0)) * dm.Ck + j;
-      const bool live = i < dm.Cq && oq[(size_t)blk * dm.Cq + i + 1] > oq[(size_t)blk * dm.Cq + i];
-      const float mu_i = live ? mu[ent] : 0.f, dS_i = live ? dS[ent] : 0.f;
-      __syncthreads();                                  // previous users of the gradient tiles are done
-      if (tid == 0) {
-        tc::mbar_expect_tx(&bar_g, 2 * kTile);
-        const int row = (int)(((size_t)pq * dm.SB + pl) * dm.Cq + i0), col = j * D;
-        tc::tma_load_2d(sm + oDka, &tm_dka, col, row, &bar_g); tc::tma_load_2d(sm + oDka + TI * 128, &tm_dka, col + 64, row, &bar_g);
-        tc::tma_load_2d(sm + oDnu, &tm_dnu, col, row, &bar_g); tc::tma_load_2d(sm + oDnu + TI * 128, &tm_dnu, col + 64, row, &bar_g);
-      }
-      if (!tc::mbar_wait(&bar_g, ph_g)) ok = false;
-      ph_g ^= 1;
-      // rows of query clusters whose segment is empty were never written: clear them
-      if (!live) {
+    if (!tc::mbar_wait(&bar_kv, ph_kv)) ok = false;
+    ph_kv ^= 1;
+    bool started = false;                                 // dK^T / dV^T accumulate in TMEM over all (i tile, plane)
+    for (int i0 = 0; i0 < dm.Cq && ok; i0 += TI) {
+      // sigma * qbar tile as bf16 hi + lo (thread = row)
+      __syncthreads();
+      {
+        const int i = i0 + tid;
+        const float* src = qbar + ((size_t)pq * dm.Cq + (i < dm.Cq ? i : 0)) * D;
 #pragma unroll
         for (int ck = 0; ck < D / 8; ++ck) {
+          uint32_t wh[4], wl[4];
+          const float4 f0 = i < dm.Cq ? ld4(src + ck * 8) : make_float4(0.f, 0.f, 0.f, 0.f);
+          const float4 f1 = i < dm.Cq ? ld4(src + ck * 8 + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+          const float x[8] = {f0.x * dm.sigma, f0.y * dm.sigma, f0.z * dm.sigma, f0.w * dm.sigma,
+                              f1.x * dm.sigma, f1.y * dm.sigma, f1.z * dm.sigma, f1.w * dm.sigma};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            __nv_bfloat162 hh = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]);
+            __nv_bfloat162 ll = __floats2bfloat162_rn(x[2 * e] - __low2float(hh), x[2 * e + 1] - __high2float(hh));
+            wh[e] = *reinterpret_cast<uint32_t*>(&hh); wl[e] = *reinterpret_cast<uint32_t*>(&ll);
+          }
           const uint32_t off = (ck >> 3) * TI * 128 + tc::sw128_off(tid, ck & 7);
-          *reinterpret_cast<uint4*>(sm + oDka + off) = make_uint4(0u, 0u, 0u, 0u);
-          *reinterpret_cast<uint4*>(sm + oDnu + off) = make_uint4(0u, 0u, 0u, 0u);
+          *reinterpret_cast<uint4*>(sm + oQhi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
+          *reinterpret_cast<uint4*>(sm + oQlo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
         }
       }
-      for (int c0 = kbeg; c0 < kend && ok; c0 += NU) {
+      for (int pl = 0; pl < dm.SB && ok; ++pl) {
+        const int kend = ok_[pl + 1];
+        if (kend <= c0) continue;                         // this plane does not see the chunk
         const int nk = min(NU, kend - c0);
-        tc::fence_async_smem();
-        __syncthreads();                                // K/V tiles and w tiles of the previous chunk are free
+        const int i = i0 + tid, blk = dm.causal ? pl + 1 : 0;
+        const size_t gent = (((size_t)pq * dm.SB + pl) * dm.Ck + j) * dm.Cq + (i < dm.Cq ? i : 0);     // gradients: [plane][j][i]
+        const size_t ent = (((size_t)pq * dm.SB + pl) * dm.Cq + (i < dm.Cq ? i : 0)) * dm.Ck + j;      // summaries: [plane][i][j]
+        const bool live = i < dm.Cq && oq[(size_t)blk * dm.Cq + i + 1] > oq[(size_t)blk * dm.Cq + i];
+        const float mu_i = live ? mu[ent] : 0.f, dS_i = live ? dS[gent] : 0.f;
+        __syncthreads();                                  // previous users of the gradient and w tiles are done
         if (tid == 0) {
-          tc::mbar_expect_tx(&bar_kv, 2 * kKeys);
-          const int row = (int)((size_t)pk * dm.N + c0);
-          tc::tma_load_2d(sm + oK, &tm_K, 0, row, &bar_kv); tc::tma_load_2d(sm + oK + NU * 128, &tm_K, 64, row, &bar_kv);
-          tc::tma_load_2d(sm + oV, &tm_V, 0, row, &bar_kv); tc::tma_load_2d(sm + oV + NU * 128, &tm_V, 64, row, &bar_kv);
-          if (!tc::mbar_wait(&bar_kv, ph_kv)) ok = false;
+          tc::mbar_expect_tx(&bar_g, 2 * kTile);
+          const int row = (int)((((size_t)pq * dm.SB + pl) * dm.Ck + j) * dm.Cq + i0);
+          tc::tma_load_2d(sm + oDka, &tm_dka, 0, row, &bar_g); tc::tma_load_2d(sm + oDka + TI * 128, &tm_dka, 64, row, &bar_g);
+          tc::tma_load_2d(sm + oDnu, &tm_dnu, 0, row, &bar_g); tc::tma_load_2d(sm + oDnu + TI * 128, &tm_dnu, 64, row, &bar_g);
+        }
+        if (!tc::mbar_wait(&bar_g, ph_g)) ok = false;
+        ph_g ^= 1;
+        // rows of query clusters whose segment is empty (or beyond Cq) were never written: clear them
+        if (!live) {
+#pragma unroll
+          for (int ck = 0; ck < D / 8; ++ck) {
+            const uint32_t off = (ck >> 3) * TI * 128 + tc::sw128_off(tid, ck & 7);
+            *reinterpret_cast<uint4*>(sm + oDka + off) = make_uint4(0u, 0u, 0u, 0u);
+            *reinterpret_cast<uint4*>(sm + oDnu + off) = make_uint4(0u, 0u, 0u, 0u);
+          }
+        }
+        tc::fence_async_smem();
+        tc::fence_before_sync();
+        __syncthreads();
+        if (tid == 0) {
           tc::fence_after_sync();
           const uint32_t idesc = tc::idesc_bf16(TI, NU, 0, 0);
 #pragma unroll
@@ -136,7 +149,6 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
                             tc::smem_desc_sw128(aV + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
           tc::mma_commit(&bar1);
         }
-        ph_kv ^= 1;
         __syncwarp();
         if (!tc::mbar_wait(&bar1, ph1)) ok = false;
         ph1 ^= 1;
@@ -171,7 +183,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
 #pragma unroll
           for (int ks = 0; ks < TI / 16; ++ks)
             tc::mma_bf16_ss(tbase + cDK, tc::smem_desc_sw128(aDka + ks * 16 * 128, TI * 128, 1024),
-                            tc::smem_desc_sw128(aW + ks * 16 * 128, TI * 128, 1024), idesc, ks > 0);
+                            tc::smem_desc_sw128(aW + ks * 16 * 128, TI * 128, 1024), idesc, started || ks > 0);
           if (dm.agg_grad) {
 #pragma unroll
             for (int ks = 0; ks < TI / 16; ++ks)
@@ -181,33 +193,35 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
 #pragma unroll
           for (int ks = 0; ks < TI / 16; ++ks)
             tc::mma_bf16_ss(tbase + cDV, tc::smem_desc_sw128(aDnu + ks * 16 * 128, TI * 128, 1024),
-                            tc::smem_desc_sw128(aW + ks * 16 * 128, TI * 128, 1024), idesc, ks > 0);
+                            tc::smem_desc_sw128(aW + ks * 16 * 128, TI * 128, 1024), idesc, started || ks > 0);
           tc::mma_commit(&bar2);
         }
+        started = true;
         __syncwarp();
         if (!tc::mbar_wait(&bar2, ph2)) ok = false;
         ph2 ^= 1;
         tc::fence_after_sync();
-        // read-out: thread = d, columns = keys of the chunk; add into the fp32 accumulators
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-          float a[32], b[32];
-          tc::tmem_ld32(tlane + cDK + 32 * hh, a);
-          tc::tmem_ld32(tlane + cDV + 32 * hh, b);
-          if (ok) {
-#pragma unroll
-            for (int u = 0; u < 32; ++u) {
-              if (32 * hh + u < nk) {
-                const size_t at = ((size_t)pq * dm.N + c0 + 32 * hh + u) * D + tid;
-                dK_perm[at] += a[u];
-                dV_perm[at] += b[u];
-              }
-            }
-          }
-        }
-        tc::fence_before_sync();
       }
     }
+    // read-out once per key chunk: thread = d, columns = keys; add into the fp32 accumulators
+    const int nkc = min(NU, kvis - c0);
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+      float a[32], b[32];
+      tc::tmem_ld32(tlane + cDK + 32 * hh, a);
+      tc::tmem_ld32(tlane + cDV + 32 * hh, b);
+      if (ok && started) {
+#pragma unroll
+        for (int u = 0; u < 32; ++u) {
+          if (32 * hh + u < nkc) {
+            const size_t at = ((size_t)pq * dm.N + c0 + 32 * hh + u) * D + tid;
+            dK_perm[at] += a[u];
+            dV_perm[at] += b[u];
+          }
+        }
+      }
+    }
+    tc::fence_before_sync();
   }
   tc::fence_before_sync();
   __syncthreads();
@@ -225,9 +239,9 @@ int summ_bwd_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* of
                 const float* mu, const void* dkappa, const void* dnu, const float* dS, float* dK_perm, float* dV_perm,
                 int* status, cudaStream_t st) {
   CUtensorMap tdka, tdnu, tK, tV;
-  const uint64_t grows = (uint64_t)d.B * d.Hq * d.SB * d.Cq, gcols = (uint64_t)d.Ck * sb::D;
-  int rc = make_tmap_bf16_pitched(&tdka, dkappa, grows, gcols, gcols * 2, sb::TI);
-  if (rc == MUSE_OK) rc = make_tmap_bf16_pitched(&tdnu, dnu, grows, gcols, gcols * 2, sb::TI);
+  const uint64_t grows = (uint64_t)d.B * d.Hq * d.SB * d.Ck * d.Cq;       // gradient entries, [plane][j][i]
+  int rc = make_tmap_bf16_rows(&tdka, dkappa, grows, sb::D, sb::TI);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tdnu, dnu, grows, sb::D, sb::TI);
   if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tK, Kp, (uint64_t)d.B * d.Hkv * d.N, sb::D, sb::NU);
   if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tV, Vp, (uint64_t)d.B * d.Hkv * d.N, sb::D, sb::NU);
   if (rc != MUSE_OK) return rc;
