@@ -585,8 +585,8 @@ k_summ_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const in
 // ---------------------------------------------------------------------------------------------
 // Final assembly
 // ---------------------------------------------------------------------------------------------
-template <class T, int D>
-__global__ void k_final_dq(Dims dm, const float* __restrict__ dQacc, const float* __restrict__ dq_part,
+template <class T, int D, class PT>      // PT: element type of the per-(query, slot) dq partials
+__global__ void k_final_dq(Dims dm, const float* __restrict__ dQacc, const PT* __restrict__ dq_part,
                            const int32_t* __restrict__ sel, int use_ret, T* __restrict__ dQ) {
   const int pq = blockIdx.y;
   const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
@@ -599,7 +599,7 @@ __global__ void k_final_dq(Dims dm, const float* __restrict__ dQacc, const float
     for (int s = 0; s < dm.m; ++s) {
       if (sel[row * dm.m + s] < 0) continue;
 #pragma unroll
-      for (int k = 0; k < D / 32; ++k) acc[k] += dq_part[(row * dm.m + s) * D + lane + 32 * k];
+      for (int k = 0; k < D / 32; ++k) acc[k] += to_f(dq_part[(row * dm.m + s) * D + lane + 32 * k]);
     }
   }
 #pragma unroll
@@ -635,7 +635,7 @@ __global__ void k_final_dkv(Dims dm, const int32_t* __restrict__ perm_k, const f
 int local_bwd_tc(const Dims& d, const void* Q, const void* K, const void* V, const void* dO, const float* LSE,
                  const float* delta, float* dQacc, float* dK_orig, float* dV_orig, int* status, cudaStream_t st);
 int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, const void* Vp, const float* LSE,
-               const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, float* dq_part,
+               const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, void* dq_part,
                float* dK_perm, float* dV_perm, int* status, cudaStream_t st);
 
 bool far_bwd_tc_supported(const Dims& d, int dtype);
@@ -769,7 +769,10 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
     MUSE_LAUNCH_OK();
   }
   prof_mark("k_final_dq", st);
-  k_final_dq<T, D><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.dQacc, w.dq_part, sel, use_ret, dQ);
+  if (kTensor)
+    k_final_dq<T, D, __nv_bfloat16><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.dQacc, (const __nv_bfloat16*)w.dq_part, sel, use_ret, dQ);
+  else
+    k_final_dq<T, D, float><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.dQacc, w.dq_part, sel, use_ret, dQ);
   MUSE_LAUNCH_OK();
   prof_mark("k_final_dkv", st);
   k_final_dkv<T, D><<<dim3(cdiv(d.N * (D / 4), 256), pk), 256, 0, st>>>(d, perm_k, w.dK_orig, w.dV_orig, w.dK_perm, w.dV_perm,

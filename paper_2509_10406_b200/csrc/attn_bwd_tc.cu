@@ -230,7 +230,7 @@ __global__ void __launch_bounds__(128)
 k_ret_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO, const bf16* __restrict__ Kp,
                 const bf16* __restrict__ Vp, const float* __restrict__ LSE, const float* __restrict__ delta,
                 const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
-                float* __restrict__ dq_part, int* __restrict__ status) {
+                bf16* __restrict__ dq_part, int* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar[2];
   __shared__ uint32_t tbase_s;
@@ -260,9 +260,25 @@ k_ret_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO
     const float L2 = tid < nq ? LSE[t] * kLog2e : 0.f, dl = tid < nq ? delta[t] : 0.f;
     const bool any = dq_rows_tc<D>(c, Kb, Vb, k0, k1, [&](int) { return k1 - 1; }, dm.sigma * kLog2e, L2, dl, tid);
     if (c.ok) {
-      float* dst = dq_part + ((size_t)pq * dm.N * dm.m + pid_s[tid]) * D;
-      if (any) read_acc_row<D>(c, 2 * kBN, dm.sigma, dst, tid < nq, tid);
-      else if (tid < nq) for (int i = 0; i < D; i += 4) *reinterpret_cast<float4*>(dst + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+      bf16* dst = dq_part + ((size_t)pq * dm.N * dm.m + pid_s[tid]) * D;       // bf16 row per (query, slot)
+      const uint32_t tq = c.tbase + ((uint32_t)((tid >> 5) * 32) << 16) + 2 * kBN;
+#pragma unroll
+      for (int d0 = 0; d0 < D; d0 += 32) {
+        float v[32];
+        if (any) tc::tmem_ld32(tq + d0, v);
+        if (tid < nq) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              __nv_bfloat162 b2 = any ? __floats2bfloat162_rn(v[i + 2 * e] * dm.sigma, v[i + 2 * e + 1] * dm.sigma) : __floats2bfloat162_rn(0.f, 0.f);
+              w[e] = *reinterpret_cast<uint32_t*>(&b2);
+            }
+            *reinterpret_cast<uint4*>(dst + d0 + i) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
     }
     tc::fence_before_sync();
   }
@@ -505,7 +521,7 @@ int local_bwd_tc(const Dims& d, const void* Q, const void* K, const void* V, con
 }
 
 int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, const void* Vp, const float* LSE,
-               const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, float* dq_part,
+               const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, void* dq_part,
                float* dK_perm, float* dV_perm, int* status, cudaStream_t st) {
   const int pq = d.B * d.Hq;
   prof_mark("k_ret_bwd_dkdv_tc", st);
@@ -513,7 +529,7 @@ int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, con
                  (const bf16*)Vp, LSE, delta, off_k, goff, pairs, dK_perm, dV_perm, status);
   prof_mark("k_ret_bwd_dq_tc", st);
   MUSE_TC_LAUNCH(k_ret_bwd_dq_tc, RowsSmem, dim3(d.Ck, d.SB * kRetSplitRows, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
-                 (const bf16*)Vp, LSE, delta, off_k, goff, pairs, dq_part, status);
+                 (const bf16*)Vp, LSE, delta, off_k, goff, pairs, (bf16*)dq_part, status);
   return MUSE_OK;
 }
 

@@ -15,7 +15,7 @@ bool far_fwd_tc_supported(const Dims& d, int dtype);
 int far_fwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const int32_t* off_q, const int32_t* perm_q,
                const int32_t* sel_in, int32_t* sel_out, float* o_far, float* lse_far, int* status, cudaStream_t st);
 int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
-               const int32_t* pairs, float* o_part, float* l_part, int* status, cudaStream_t st);
+               const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st);
 
 // plane of a query = index of the accumulated-summary plane it reads: block - 1 when causal
 // (block 0 sees no far field), 0 when non-causal.
@@ -25,28 +25,41 @@ __device__ __forceinline__ int query_plane(const Dims& d, int t) { return d.caus
 // Inverse index for retrieval (Section "Exact retrieval": "an inverse index mapping each
 // (cluster, block) to the queries that retrieve it").  Group key = plane * Ck + cluster.
 // ---------------------------------------------------------------------------------------------
+// Thread e handles (slot = e / N, query = e % N): the lanes of a warp are consecutive queries,
+// which often retrieve the same cluster in the same slot, so equal keys are combined with a warp
+// match and only one atomic per distinct key and warp reaches memory.
 __global__ void k_ret_count(Dims d, const int32_t* __restrict__ sel, int32_t* __restrict__ cnt) {
   const int pq = blockIdx.y;
   const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= (long long)d.N * d.m) return;
-  const int t = (int)(e / d.m);
-  const int c = sel[(size_t)pq * d.N * d.m + e];
-  const int pl = query_plane(d, t);
-  if (c >= 0 && pl >= 0) atomicAdd(&cnt[(size_t)pq * d.SB * d.Ck + (size_t)pl * d.Ck + c], 1);
+  int key = -1;
+  if (e < (long long)d.N * d.m) {
+    const int t = (int)(e % d.N), k = (int)(e / d.N);
+    const int c = sel[((size_t)pq * d.N + t) * d.m + k];
+    const int pl = query_plane(d, t);
+    if (c >= 0 && pl >= 0) key = pl * d.Ck + c;
+  }
+  const unsigned peers = __match_any_sync(0xffffffffu, key);
+  const int lane = threadIdx.x & 31;
+  if (key >= 0 && lane == __ffs(peers) - 1) atomicAdd(&cnt[(size_t)pq * d.SB * d.Ck + key], __popc(peers));
 }
 
 __global__ void k_ret_fill(Dims d, const int32_t* __restrict__ sel, int32_t* __restrict__ cursor,
                            int32_t* __restrict__ pairs) {
   const int pq = blockIdx.y;
   const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= (long long)d.N * d.m) return;
-  const int t = (int)(e / d.m);
-  const int c = sel[(size_t)pq * d.N * d.m + e];
-  const int pl = query_plane(d, t);
-  if (c >= 0 && pl >= 0) {
-    int pos = atomicAdd(&cursor[(size_t)pq * d.SB * d.Ck + (size_t)pl * d.Ck + c], 1);
-    pairs[(size_t)pq * d.N * d.m + pos] = (int)e;
+  int key = -1, pid = 0;
+  if (e < (long long)d.N * d.m) {
+    const int t = (int)(e % d.N), k = (int)(e / d.N);
+    const int c = sel[((size_t)pq * d.N + t) * d.m + k];
+    const int pl = query_plane(d, t);
+    if (c >= 0 && pl >= 0) { key = pl * d.Ck + c; pid = t * d.m + k; }
   }
+  const unsigned peers = __match_any_sync(0xffffffffu, key);
+  const int lane = threadIdx.x & 31, leader = __ffs(peers) - 1;
+  int base = 0;
+  if (key >= 0 && lane == leader) base = atomicAdd(&cursor[(size_t)pq * d.SB * d.Ck + key], __popc(peers));
+  base = __shfl_sync(0xffffffffu, base, leader);
+  if (key >= 0) pairs[(size_t)pq * d.N * d.m + base + __popc(peers & ((1u << lane) - 1u))] = pid;
 }
 
 size_t ret_index_elems(const Dims& d) {
@@ -426,10 +439,10 @@ k_local_fwd(Dims dm, const T* __restrict__ Q, const T* __restrict__ K, const T* 
 // ---------------------------------------------------------------------------------------------
 // Merge: L = LSE over components, O = sum_c exp(lse_c - L) o_c.  One warp per query.
 // ---------------------------------------------------------------------------------------------
-template <class T, int D>
+template <class T, int D, class PT>      // PT: element type of the retrieval partial outputs
 __global__ void k_merge(Dims dm, const float* __restrict__ o_far, const float* __restrict__ lse_far,
                         const float* __restrict__ o_loc, const float* __restrict__ lse_loc,
-                        const float* __restrict__ o_part, const float* __restrict__ l_part,
+                        const PT* __restrict__ o_part, const float* __restrict__ l_part,
                         const int32_t* __restrict__ sel, T* __restrict__ O, float* __restrict__ LSE) {
   const int pq = blockIdx.y;
   const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
@@ -472,7 +485,7 @@ __global__ void k_merge(Dims dm, const float* __restrict__ o_far, const float* _
     if (lp == -INFINITY) continue;
     const float w = expf(lp - mx);
 #pragma unroll
-    for (int k = 0; k < D / 32; ++k) acc[k] = fmaf(w, o_part[(row * m + s) * D + lane + 32 * k], acc[k]);
+    for (int k = 0; k < D / 32; ++k) acc[k] = fmaf(w, to_f(o_part[(row * m + s) * D + lane + 32 * k]), acc[k]);
   }
 #pragma unroll
   for (int k = 0; k < D / 32; ++k) O[row * D + lane + 32 * k] = from_f<T>(acc[k] * inv);
@@ -559,7 +572,11 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
     }
   }
   prof_mark("k_merge", st);
-  k_merge<T, D><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.o_far, w.lse_far, w.o_loc, w.lse_loc, w.o_part, w.l_part, sel, O, LSE);
+  if (kTensor)
+    k_merge<T, D, __nv_bfloat16><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.o_far, w.lse_far, w.o_loc, w.lse_loc,
+                                                                       (const __nv_bfloat16*)w.o_part, w.l_part, sel, O, LSE);
+  else
+    k_merge<T, D, float><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.o_far, w.lse_far, w.o_loc, w.lse_loc, w.o_part, w.l_part, sel, O, LSE);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }

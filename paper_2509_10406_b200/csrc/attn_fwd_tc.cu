@@ -209,7 +209,7 @@ template <int D>
 __global__ void __launch_bounds__(128)
 k_ret_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, const bf16* __restrict__ Vp,
              const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
-             float* __restrict__ o_part, float* __restrict__ l_part, int* __restrict__ status) {
+             bf16* __restrict__ o_part, float* __restrict__ l_part, int* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar[2];
   __shared__ uint32_t tbase_s;
@@ -243,9 +243,17 @@ k_ret_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, c
     if (c.ok && tid < nq) {
       const size_t pid = (size_t)pq * dm.N * dm.m + pid_s[tid];
       const float inv = l > 0.f ? 1.f / l : 0.f;
-      float4* dst = reinterpret_cast<float4*>(o_part + pid * D);
+      uint4* dst = reinterpret_cast<uint4*>(o_part + pid * D);          // normalised partial output, bf16 row
 #pragma unroll
-      for (int i = 0; i < D / 4; ++i) dst[i] = make_float4(o[4 * i] * inv, o[4 * i + 1] * inv, o[4 * i + 2] * inv, o[4 * i + 3] * inv);
+      for (int i = 0; i < D / 8; ++i) {
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          __nv_bfloat162 b2 = __floats2bfloat162_rn(o[8 * i + 2 * e] * inv, o[8 * i + 2 * e + 1] * inv);
+          w[e] = *reinterpret_cast<uint32_t*>(&b2);
+        }
+        dst[i] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
       l_part[pid] = l > 0.f ? (m2 + log2f(l)) * 0.6931471805599453f : -INFINITY;
     }
   }
@@ -269,15 +277,15 @@ int local_fwd_tc(const Dims& d, const void* Q, const void* K, const void* V, flo
 }
 
 int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
-               const int32_t* pairs, float* o_part, float* l_part, int* status, cudaStream_t st) {
+               const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st) {
   dim3 grid(d.Ck, d.SB * kRetFwdSplit, d.B * d.Hq);
   prof_mark("k_ret_fwd_tc", st);
   if (d.D == 128) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdTcSmem<128>::total));
-    k_ret_fwd_tc<128><<<grid, 128, FwdTcSmem<128>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs, o_part, l_part, status);
+    k_ret_fwd_tc<128><<<grid, 128, FwdTcSmem<128>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs, (bf16*)o_part, l_part, status);
   } else {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdTcSmem<64>::total));
-    k_ret_fwd_tc<64><<<grid, 128, FwdTcSmem<64>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs, o_part, l_part, status);
+    k_ret_fwd_tc<64><<<grid, 128, FwdTcSmem<64>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs, (bf16*)o_part, l_part, status);
   }
   MUSE_LAUNCH_OK();
   return MUSE_OK;
