@@ -324,15 +324,24 @@ __device__ __forceinline__ void dkdv_step_tc(BwdCtx& c, const float* __restrict_
   float p[kBN], g[kBN];
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
-    float s[32], dp[32];
+    float s[32], dp[32], Lc[32], dc[32];
     tc::tmem_ld32(t_s + 32 * h, s);
     tc::tmem_ld32(t_dp + 32 * h, dp);
+    // the per-column L and delta come out of shared memory in vector loads before the loop: with
+    // one or two warps per scheduler a load inside each iteration would expose its latency 64 times
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float4 a = *reinterpret_cast<const float4*>(Ls + 32 * h + 4 * k), b = *reinterpret_cast<const float4*>(ds + 32 * h + 4 * k);
+      Lc[4 * k] = a.x; Lc[4 * k + 1] = a.y; Lc[4 * k + 2] = a.z; Lc[4 * k + 3] = a.w;
+      dc[4 * k] = b.x; dc[4 * k + 1] = b.y; dc[4 * k + 2] = b.z; dc[4 * k + 3] = b.w;
+    }
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
       const int col = 32 * h + i;
-      const float pv = mask(col) ? exp2f(s[i] * scale2 - Ls[col]) : 0.f;
+      const float e = exp2f(s[i] * scale2 - Lc[i]);
+      const float pv = mask(col) ? e : 0.f;
       p[col] = pv;
-      g[col] = pv * (dp[i] - ds[col]);
+      g[col] = pv * (dp[i] - dc[i]);
     }
   }
   store_row64(c.sm + SM::pt, tid, p);
@@ -366,7 +375,7 @@ k_local_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict_
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar[2];
   __shared__ uint32_t tbase_s;
-  __shared__ float Ls[kBN], ds[kBN];
+  __shared__ __align__(16) float Ls[kBN], ds[kBN];
   const int tid = threadIdx.x;
   BwdCtx c;
   bwd_setup(c, sm_raw, bar, &tbase_s, SM::cols, tid);
@@ -440,7 +449,7 @@ k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar[2];
   __shared__ uint32_t tbase_s;
-  __shared__ float Ls[kBN], ds[kBN];
+  __shared__ __align__(16) float Ls[kBN], ds[kBN];
   __shared__ int32_t tok_s[kBN];
   const int tid = threadIdx.x;
   const int j = blockIdx.x, pl = blockIdx.y / kRetSplit, sub = blockIdx.y % kRetSplit, pq = blockIdx.z;

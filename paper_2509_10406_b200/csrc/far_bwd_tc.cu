@@ -28,6 +28,12 @@ constexpr uint32_t cS = 0, cDP = 64, cDNU = 128, cDKA = 256, cDQ = 384;   // TME
 constexpr float kLog2e = 1.4426950408889634f;
 }  // namespace fb
 
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __global__ void __launch_bounds__(fb::THREADS, 1)
 k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_constant__ CUtensorMap tm_klo,
              const __grid_constant__ CUtensorMap tm_nu, const bf16* __restrict__ Q, const bf16* __restrict__ dO,
@@ -40,7 +46,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   __shared__ uint64_t bar_full, bar1, bar2;
   __shared__ uint32_t tbase_s;
   __shared__ int32_t rows[NP * NR];
-  __shared__ float Ls[NP * NR], ds[NP * NR], qb[D], part[2][TJ], dots[2][TJ];
+  __shared__ __align__(16) float Ls[NP * NR], ds[NP * NR], qb[D], part[2][TJ], dots[2][TJ];
   const int i = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z;
   const int blk = dm.causal ? pl + 1 : 0, Ck = dm.Ck, NJ = Ck / TJ, MW = Ck >> 5, m = dm.m;
   const int tid = threadIdx.x, warp = tid >> 5, wg = tid >> 7, L = tid & 127;
@@ -90,21 +96,36 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     for (int e = tid; e < ns * m; e += THREADS) {
       const int r = e / m, k = e % m;
       const int c = sel[((size_t)pq * dm.N + rows[r]) * m + k];
-      if (c >= 0 && c < Ck) atomicOr(&smask[r * MW + (c >> 5)], 1u << (c & 31));
+      if (c >= 0 && c < Ck) atomicOr(&smask[(c >> 5) * (NP * NR) + r], 1u << (c & 31));     // [word][row]
     }
     tc::fence_async_smem();
     __syncthreads();
 
+#ifdef MUSE_PHASE_CLOCKS
+    long long pc[6] = {0, 0, 0, 0, 0, 0};
+#endif
+    float bnext = beta[ent0 + L];
     for (int jt = 0; jt < NJ && ok; ++jt) {
       const int j = jt * TJ + L;
+#ifdef MUSE_PHASE_CLOCKS
+      long long k0_ = clock64(), k1_ = 0, k2_ = 0, k3_ = 0, k4_ = 0;
+#endif
       if (tid == 0) {
         tc::mbar_expect_tx(&bar_full, 3 * kTile);
         const int row = (int)(ent0 + (size_t)jt * TJ);
         tc::tma_load_2d(sm + oHi, &tm_khi, 0, row, &bar_full); tc::tma_load_2d(sm + oHi + TJ * 128, &tm_khi, 64, row, &bar_full);
         tc::tma_load_2d(sm + oLo, &tm_klo, 0, row, &bar_full); tc::tma_load_2d(sm + oLo + TJ * 128, &tm_klo, 64, row, &bar_full);
         tc::tma_load_2d(sm + oNu, &tm_nu, 0, row, &bar_full); tc::tma_load_2d(sm + oNu + TJ * 128, &tm_nu, 64, row, &bar_full);
+        if (jt + 1 < NJ) {                    // start pulling the next cluster tile into L2 while this one is processed
+          const int nrow = row + TJ;
+          tc::tma_prefetch_2d(&tm_khi, 0, nrow); tc::tma_prefetch_2d(&tm_khi, 64, nrow);
+          tc::tma_prefetch_2d(&tm_klo, 0, nrow); tc::tma_prefetch_2d(&tm_klo, 64, nrow);
+          tc::tma_prefetch_2d(&tm_nu, 0, nrow); tc::tma_prefetch_2d(&tm_nu, 64, nrow);
+        }
       }
-      const float bj = beta[ent0 + j];
+      const float bj = bnext;                               // loaded one tile ahead
+      const float sig2 = dm.sigma * kLog2e, bj2 = bj * kLog2e;
+      if (jt + 1 < NJ) bnext = beta[ent0 + j + TJ];
       float gsum = 0.f;
       for (int p = 0; p < np && ok; ++p) {
         const uint32_t aQ = tc::smem_u32(sm + oQ + p * kRows), aDO = tc::smem_u32(sm + oDO + p * kRows);
@@ -130,32 +151,57 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
         if (!tc::mbar_wait(&bar1, ph1)) ok = false;
         ph1 ^= 1;
         tc::fence_after_sync();
+#ifdef MUSE_PHASE_CLOCKS
+        if (p == 0) k1_ = clock64();
+#endif
         {
           float s[32], dp[32];
           tc::tmem_ld32(tlane + cS + 32 * wg, s);
           tc::tmem_ld32(tlane + cDP + 32 * wg, dp);
+#ifdef MUSE_PHASE_CLOCKS
+          if (p == 0 && tid == 0 && blockIdx.x == 5 && blockIdx.y == 3 && blockIdx.z == 0 && jt == 3) status[32] = (int)(clock64() - k1_);
+#endif
           uint32_t pw[16], gw[16];
+          // per-row L, delta and retrieved-cluster bits: vector loads ahead of the arithmetic loop
+          float Lc[32], dc[32];
+          uint32_t mk[32];
+          const int rb = p * NR + 32 * wg;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            const float4 a = *reinterpret_cast<const float4*>(Ls + rb + 4 * k), b = *reinterpret_cast<const float4*>(ds + rb + 4 * k);
+            const uint4 w = *reinterpret_cast<const uint4*>(smask + (j >> 5) * (NP * NR) + rb + 4 * k);
+            Lc[4 * k] = a.x; Lc[4 * k + 1] = a.y; Lc[4 * k + 2] = a.z; Lc[4 * k + 3] = a.w;
+            dc[4 * k] = b.x; dc[4 * k + 1] = b.y; dc[4 * k + 2] = b.z; dc[4 * k + 3] = b.w;
+            mk[4 * k] = w.x; mk[4 * k + 1] = w.y; mk[4 * k + 2] = w.z; mk[4 * k + 3] = w.w;
+          }
+          const bool alive = bj != -INFINITY;
 #pragma unroll
           for (int c = 0; c < 32; c += 2) {
             float pv[2], gv[2];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-              const int r = p * NR + 32 * wg + c + h;
-              const bool far = bj != -INFINITY && r < ns && !((smask[r * MW + (j >> 5)] >> (j & 31)) & 1u);
-              pv[h] = far ? exp2f(fmaf(s[c + h], dm.sigma, bj) * kLog2e - Ls[r]) : 0.f;
-              gv[h] = pv[h] * (dp[c + h] - ds[r]);
+              const bool far = alive && rb + c + h < ns && !((mk[c + h] >> (j & 31)) & 1u);
+              const float e = fast_exp2(fmaf(s[c + h], sig2, bj2) - Lc[c + h]);
+              pv[h] = far ? e : 0.f;
+              gv[h] = pv[h] * (dp[c + h] - dc[c + h]);
               gsum += gv[h];
             }
             __nv_bfloat162 a = __floats2bfloat162_rn(pv[0], pv[1]), b = __floats2bfloat162_rn(gv[0], gv[1]);
             pw[c >> 1] = *reinterpret_cast<uint32_t*>(&a);
             gw[c >> 1] = *reinterpret_cast<uint32_t*>(&b);
           }
+#ifdef MUSE_PHASE_CLOCKS
+          if (p == 0 && tid == 0 && blockIdx.x == 5 && blockIdx.y == 3 && blockIdx.z == 0 && jt == 3) status[33] = (int)(clock64() - k1_);
+#endif
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
             *reinterpret_cast<uint4*>(sm + oPt + tc::sw128_off(L, 4 * wg + ch)) = make_uint4(pw[4 * ch], pw[4 * ch + 1], pw[4 * ch + 2], pw[4 * ch + 3]);
             *reinterpret_cast<uint4*>(sm + oGt + tc::sw128_off(L, 4 * wg + ch)) = make_uint4(gw[4 * ch], gw[4 * ch + 1], gw[4 * ch + 2], gw[4 * ch + 3]);
           }
         }
+#ifdef MUSE_PHASE_CLOCKS
+        if (p == 0) k2_ = clock64();
+#endif
         tc::fence_async_smem();
         tc::fence_before_sync();
         __syncthreads();
@@ -187,6 +233,9 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
         tc::fence_after_sync();
       }
       ph_full ^= 1;
+#ifdef MUSE_PHASE_CLOCKS
+      k3_ = clock64();
+#endif
       // ---- tile read-out: warpgroup 0 -> dnu, warpgroup 1 -> dkappa; both need sum_r g
       part[wg][L] = gsum;
       __syncthreads();
@@ -200,37 +249,63 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       for (int d0 = 0; d0 < D; d0 += 32) {
         float v[32];
         tc::tmem_ld32(tlane + (wg == 0 ? cDNU : cDKA) + d0, v);
+        // operands of this 32-wide slice first (vector loads), arithmetic after
+        float qv[32];
+        uint4 ra[4], rb[4];
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           const int d = d0 + 8 * ch, kb = d >> 6, c = (d & 63) >> 3;
           const uint32_t off = kb * TJ * 128 + tc::sw128_off(L, c);
+          ra[ch] = *reinterpret_cast<const uint4*>(sm + (wg == 0 ? oNu : oHi) + off);
+          rb[ch] = wg == 0 ? make_uint4(0u, 0u, 0u, 0u) : *reinterpret_cast<const uint4*>(sm + oLo + off);
+          const float4 q0 = *reinterpret_cast<const float4*>(qb + d), q1 = *reinterpret_cast<const float4*>(qb + d + 4);
+          qv[8 * ch] = q0.x; qv[8 * ch + 1] = q0.y; qv[8 * ch + 2] = q0.z; qv[8 * ch + 3] = q0.w;
+          qv[8 * ch + 4] = q1.x; qv[8 * ch + 5] = q1.y; qv[8 * ch + 6] = q1.z; qv[8 * ch + 7] = q1.w;
+        }
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+          const int d = d0 + 8 * ch;
           float x[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e)      // rounded to the stored bf16 value so that dS matches what the key-side pass reads
-            x[e] = __bfloat162float(__float2bfloat16_rn(wg == 0 ? v[8 * ch + e] : dm.sigma * (v[8 * ch + e] - gtot * qb[d + e])));
-          uint4 ra = *reinterpret_cast<const uint4*>(sm + (wg == 0 ? oNu : oHi) + off);
-          const bf16* ha = reinterpret_cast<const bf16*>(&ra);
-          if (wg == 0) {
+            x[e] = __bfloat162float(__float2bfloat16_rn(wg == 0 ? v[8 * ch + e] : dm.sigma * (v[8 * ch + e] - gtot * qv[8 * ch + e])));
+          const bf16* ha = reinterpret_cast<const bf16*>(&ra[ch]);
+          const bf16* hb = reinterpret_cast<const bf16*>(&rb[ch]);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) dot = fmaf(x[e], __bfloat162float(ha[e]), dot);
-          } else {
-            uint4 rb = *reinterpret_cast<const uint4*>(sm + oLo + off);
-            const bf16* hb = reinterpret_cast<const bf16*>(&rb);
-#pragma unroll
-            for (int e = 0; e < 8; ++e) dot = fmaf(x[e], __bfloat162float(ha[e]) + __bfloat162float(hb[e]), dot);
-          }
+          for (int e = 0; e < 8; ++e) dot = fmaf(x[e], __bfloat162float(ha[e]) + __bfloat162float(hb[e]), dot);
           uint32_t w[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) { __nv_bfloat162 b2 = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]); w[e] = *reinterpret_cast<uint32_t*>(&b2); }
-          if (ok) *reinterpret_cast<uint4*>(dst + d) = make_uint4(w[0], w[1], w[2], w[3]);
+          // back into this thread's own row of the (now consumed) nu / kappa_hi tile; the rows leave
+          // through a cooperative, fully coalesced copy below instead of 16-byte scattered stores
+          const int kb = d >> 6, c = (d & 63) >> 3;
+          *reinterpret_cast<uint4*>(sm + (wg == 0 ? oNu : oHi) + kb * TJ * 128 + tc::sw128_off(L, c)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
+      (void)dst;
       dots[wg][L] = dot;
-      tc::fence_async_smem();          // generic reads of the tiles are ordered before the next TMA writes
+      __syncthreads();
+      if (ok) {
+        for (int e = tid; e < 2 * TJ * (D / 8); e += THREADS) {
+          const int arr = e / (TJ * (D / 8)), r = (e / (D / 8)) % TJ, ch = e % (D / 8);
+          const size_t ge = grad_by_key_cluster ? (((size_t)pq * dm.SB + pl) * Ck + jt * TJ + r) * dm.Cq + i : ent0 + (size_t)jt * TJ + r;
+          const uint4 val = *reinterpret_cast<const uint4*>(sm + (arr == 0 ? oNu : oHi) + (ch >> 3) * TJ * 128 + tc::sw128_off(r, ch & 7));
+          *reinterpret_cast<uint4*>((arr == 0 ? dnu : dkappa) + ge * D + ch * 8) = val;
+        }
+      }
+      tc::fence_async_smem();          // generic accesses to the tiles are ordered before the next TMA writes
       tc::fence_before_sync();
       __syncthreads();
       if (wg == 0 && ok) dS[gent] = gtot - dots[0][L] - dots[1][L];
+#ifdef MUSE_PHASE_CLOCKS
+      k4_ = clock64();
+      pc[0] += k1_ - k0_; pc[1] += k2_ - k1_; pc[2] += k3_ - k2_; pc[3] += k4_ - k3_; pc[4] += 1; pc[5] = np;
+#endif
     }
+#ifdef MUSE_PHASE_CLOCKS
+    if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 3 && blockIdx.z == 0 && s0 == p0)
+      for (int k = 0; k < 6; ++k) status[24 + k] = (int)pc[k];
+#endif
     // ---- dq: warpgroup p reads pass p (thread = output dim), adds into the fp32 accumulator
     for (int p = wg; p < np; p += 2) {
 #pragma unroll

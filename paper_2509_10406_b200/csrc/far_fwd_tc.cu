@@ -143,11 +143,17 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     ck1 = clock64();
 #endif
     // ---- B: TMEM -> sc[r][j]
-    for (int jt = warp >> 2; jt < NJ; jt += kFarTcThreads / 128) {
+    float bq[2];                                        // beta of this thread's clusters, loaded ahead of the TMEM reads
+#pragma unroll
+    for (int k = 0; k < 2; ++k) { const int jt = (warp >> 2) + 4 * k; bq[k] = jt < NJ ? bep[jt * kFJ + (tid & 127)] : 0.f; }
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+      const int jt = (warp >> 2) + 4 * k;
+      if (jt >= NJ) break;
       float v[32];
       tc::tmem_ld32(tbase + ((uint32_t)((warp & 3) * 32) << 16) + jt * kFR, v);
       const int j = jt * kFJ + (tid & 127);
-      const float b = bep[j];
+      const float b = bq[k];
 #pragma unroll
       for (int r = 0; r < kFR; ++r) sc[r * Ck + j] = b == -INFINITY ? -INFINITY : fmaf(v[r], dm.sigma, b);
     }
