@@ -17,10 +17,10 @@ typedef __nv_bfloat16 bf16;
 constexpr int kBM = 128, kBN = 64;
 constexpr float kLog2e = 1.4426950408889634f;
 
-template <int D, int ROWS, class RowPtr>
+template <int D, int ROWS, int NT = 128, class RowPtr>
 __device__ __forceinline__ void fill_tile(unsigned char* dst, int n, RowPtr row_ptr, int tid) {
   constexpr int CPR = D / 8;
-  for (int e = tid; e < ROWS * CPR; e += 128) {
+  for (int e = tid; e < ROWS * CPR; e += NT) {
     const int r = e / CPR, ck = e % CPR, kb = ck >> 3, c = ck & 7;
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (r < n) v = reinterpret_cast<const uint4*>(row_ptr(r))[ck];
@@ -30,22 +30,22 @@ __device__ __forceinline__ void fill_tile(unsigned char* dst, int n, RowPtr row_
 
 // A [ROWS][D] tile held in registers between its global loads and its shared-memory stores, so
 // that the loads of the next tile are in flight while the tensor core works on the current one.
-template <int D, int ROWS> struct TileRegs { static constexpr int N = ROWS * (D / 8) / 128; uint4 v[N]; };
-template <int D, int ROWS, class RowPtr>
-__device__ __forceinline__ void tile_ldg(TileRegs<D, ROWS>& t, int n, RowPtr row_ptr, int tid) {
+template <int D, int ROWS, int NT = 128> struct TileRegs { static constexpr int N = ROWS * (D / 8) / NT; uint4 v[N]; };
+template <int D, int ROWS, int NT = 128, class RowPtr>
+__device__ __forceinline__ void tile_ldg(TileRegs<D, ROWS, NT>& t, int n, RowPtr row_ptr, int tid) {
   constexpr int CPR = D / 8;
 #pragma unroll
-  for (int k = 0; k < TileRegs<D, ROWS>::N; ++k) {
-    const int e = tid + 128 * k, r = e / CPR, ck = e % CPR;
+  for (int k = 0; k < TileRegs<D, ROWS, NT>::N; ++k) {
+    const int e = tid + NT * k, r = e / CPR, ck = e % CPR;
     t.v[k] = r < n ? __ldg(reinterpret_cast<const uint4*>(row_ptr(r)) + ck) : make_uint4(0u, 0u, 0u, 0u);
   }
 }
-template <int D, int ROWS>
-__device__ __forceinline__ void tile_sts(const TileRegs<D, ROWS>& t, unsigned char* dst, int tid) {
+template <int D, int ROWS, int NT = 128>
+__device__ __forceinline__ void tile_sts(const TileRegs<D, ROWS, NT>& t, unsigned char* dst, int tid) {
   constexpr int CPR = D / 8;
 #pragma unroll
-  for (int k = 0; k < TileRegs<D, ROWS>::N; ++k) {
-    const int e = tid + 128 * k, r = e / CPR, ck = e % CPR;
+  for (int k = 0; k < TileRegs<D, ROWS, NT>::N; ++k) {
+    const int e = tid + NT * k, r = e / CPR, ck = e % CPR;
     *reinterpret_cast<uint4*>(dst + (ck >> 3) * ROWS * 128 + tc::sw128_off(r, ck & 7)) = t.v[k];
   }
 }
@@ -60,6 +60,9 @@ template <int ROWS> __device__ __forceinline__ uint64_t desc_mn(uint32_t base, i
 }
 
 struct BwdCtx {
+#ifdef MUSE_PHASE_CLOCKS
+  long long pc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#endif
   unsigned char* sm;
   uint64_t* bar;
   uint32_t tbase, ph0, ph1;
@@ -93,6 +96,20 @@ __device__ __forceinline__ void store_row64(unsigned char* tile, int row, const 
       w[k] = *reinterpret_cast<uint32_t*>(&b);
     }
     *reinterpret_cast<uint4*>(tile + tc::sw128_off(row, ch)) = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
+// half a row (32 columns, chunks 4*half .. 4*half+3) of a [128][64] bf16 tile
+__device__ __forceinline__ void store_row32(unsigned char* tile, int row, int half, const float (&x)[32]) {
+#pragma unroll
+  for (int ch = 0; ch < 4; ++ch) {
+    uint32_t w[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      __nv_bfloat162 b = __floats2bfloat162_rn(x[ch * 8 + 2 * k], x[ch * 8 + 2 * k + 1]);
+      w[k] = *reinterpret_cast<uint32_t*>(&b);
+    }
+    *reinterpret_cast<uint4*>(tile + tc::sw128_off(row, 4 * half + ch)) = make_uint4(w[0], w[1], w[2], w[3]);
   }
 }
 
@@ -154,7 +171,7 @@ __device__ __forceinline__ bool dq_rows_tc(BwdCtx& c, const bf16* __restrict__ K
       tc::tmem_ld32(t_dp + 32 * h, dp);
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        const float p = (32 * h + i) < vis ? exp2f(s[i] * scale2 - L2) : 0.f;
+        const float p = (32 * h + i) < vis ? tc::fast_exp2(s[i] * scale2 - L2) : 0.f;
         g[32 * h + i] = p * (dp[i] - delta);
       }
     }
@@ -183,7 +200,7 @@ __device__ __forceinline__ bool dq_rows_tc(BwdCtx& c, const bf16* __restrict__ K
 // must call this; only the global store is predicated.
 template <int D>
 __device__ __forceinline__ void read_acc_row(const BwdCtx& c, uint32_t col, float f, float* __restrict__ dst, bool write, int tid) {
-  const uint32_t t = c.tbase + ((uint32_t)((tid >> 5) * 32) << 16) + col;
+  const uint32_t t = c.tbase + ((uint32_t)(((tid >> 5) & 3) * 32) << 16) + col;
 #pragma unroll
   for (int d0 = 0; d0 < D; d0 += 32) {
     float v[32];
@@ -301,13 +318,19 @@ template <int D, class Mask, class Prefetch>
 __device__ __forceinline__ void dkdv_step_tc(BwdCtx& c, const float* __restrict__ Ls, const float* __restrict__ ds,
                                              Mask mask, float scale2, bool& started, int tid, Prefetch prefetch) {
   typedef KeysSmem<D> SM;
-  const int warp = tid >> 5;
-  const uint32_t t_s = c.tbase + ((uint32_t)(warp * 32) << 16), t_dp = t_s + kBN;
+  const int warp = tid >> 5, wg = tid >> 7, row = tid & 127;       // 256 threads: warpgroup wg owns columns [32 wg, 32 wg + 32)
+  const uint32_t t_s = c.tbase + ((uint32_t)((warp & 3) * 32) << 16), t_dp = t_s + kBN;
   const uint32_t ka = tc::smem_u32(c.sm + SM::k), va = tc::smem_u32(c.sm + SM::v), qa = tc::smem_u32(c.sm + SM::q),
                  da = tc::smem_u32(c.sm + SM::dO), pa = tc::smem_u32(c.sm + SM::pt), ga = tc::smem_u32(c.sm + SM::gt);
+#ifdef MUSE_PHASE_CLOCKS
+  const long long z0 = clock64();
+#endif
   tc::fence_async_smem();
   tc::fence_before_sync();
   __syncthreads();
+#ifdef MUSE_PHASE_CLOCKS
+  const long long z1 = clock64();
+#endif
   if (tid == 0) {
     tc::fence_after_sync();
     const uint32_t idesc = tc::idesc_bf16(kBM, kBN, 0, 0);
@@ -318,17 +341,22 @@ __device__ __forceinline__ void dkdv_step_tc(BwdCtx& c, const float* __restrict_
     tc::mma_commit(&c.bar[0]);
   }
   prefetch();                                  // global loads of the next query tile, overlapped with the MMAs
+#ifdef MUSE_PHASE_CLOCKS
+  const long long z2 = clock64();
+#endif
   if (!tc::mbar_wait(&c.bar[0], c.ph0)) { c.ok = false; return; }
   c.ph0 ^= 1;
   tc::fence_after_sync();
-  float p[kBN], g[kBN];
-#pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    float s[32], dp[32], Lc[32], dc[32];
+#ifdef MUSE_PHASE_CLOCKS
+  const long long z3 = clock64();
+#endif
+  {
+    const int h = wg;
+    float s[32], dp[32], Lc[32], dc[32], p[32], g[32];
     tc::tmem_ld32(t_s + 32 * h, s);
     tc::tmem_ld32(t_dp + 32 * h, dp);
     // the per-column L and delta come out of shared memory in vector loads before the loop: with
-    // one or two warps per scheduler a load inside each iteration would expose its latency 64 times
+    // one or two warps per scheduler a load inside each iteration would expose its latency every time
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
       const float4 a = *reinterpret_cast<const float4*>(Ls + 32 * h + 4 * k), b = *reinterpret_cast<const float4*>(ds + 32 * h + 4 * k);
@@ -337,15 +365,17 @@ __device__ __forceinline__ void dkdv_step_tc(BwdCtx& c, const float* __restrict_
     }
 #pragma unroll
     for (int i = 0; i < 32; ++i) {
-      const int col = 32 * h + i;
-      const float e = exp2f(s[i] * scale2 - Lc[i]);
-      const float pv = mask(col) ? e : 0.f;
-      p[col] = pv;
-      g[col] = pv * (dp[i] - dc[i]);
+      const float e = tc::fast_exp2(s[i] * scale2 - Lc[i]);
+      const float pv = mask(32 * h + i) ? e : 0.f;
+      p[i] = pv;
+      g[i] = pv * (dp[i] - dc[i]);
     }
+    store_row32(c.sm + SM::pt, row, h, p);
+    store_row32(c.sm + SM::gt, row, h, g);
   }
-  store_row64(c.sm + SM::pt, tid, p);
-  store_row64(c.sm + SM::gt, tid, g);
+#ifdef MUSE_PHASE_CLOCKS
+  const long long z4 = clock64();
+#endif
   tc::fence_async_smem();
   tc::fence_before_sync();
   __syncthreads();
@@ -364,10 +394,16 @@ __device__ __forceinline__ void dkdv_step_tc(BwdCtx& c, const float* __restrict_
   if (!tc::mbar_wait(&c.bar[1], c.ph1)) { c.ok = false; return; }
   c.ph1 ^= 1;
   tc::fence_after_sync();
+#ifdef MUSE_PHASE_CLOCKS
+  const long long z5 = clock64();
+  c.pc[0] += z1 - z0; c.pc[1] += z2 - z1; c.pc[2] += z3 - z2; c.pc[3] += z4 - z3; c.pc[4] += z5 - z4; c.pc[5] += 1;
+#endif
 }
 
+constexpr int kKeysThreads = 256;       // keys-on-M kernels: two warpgroups share the 64 query columns
+
 template <int D>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kKeysThreads)
 k_local_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ K, const bf16* __restrict__ V,
                     const bf16* __restrict__ dO, const float* __restrict__ LSE, const float* __restrict__ delta,
                     float* __restrict__ dK_orig, float* __restrict__ dV_orig, int* __restrict__ status) {
@@ -376,7 +412,7 @@ k_local_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict_
   __shared__ uint64_t bar[2];
   __shared__ uint32_t tbase_s;
   __shared__ __align__(16) float Ls[kBN], ds[kBN];
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, row = tid & 127, wg = tid >> 7;
   BwdCtx c;
   bwd_setup(c, sm_raw, bar, &tbase_s, SM::cols, tid);
   const int tpb = cdiv(dm.Bs, kBM);
@@ -386,16 +422,16 @@ k_local_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict_
   const int k0 = bstart + kt * kBM, nk = min(kBM, bend - k0);
   const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
   const bf16* Kb = K + (size_t)pk * dm.N * D; const bf16* Vb = V + (size_t)pk * dm.N * D;
-  fill_tile<D, kBM>(c.sm + SM::k, nk, [&](int r) { return Kb + (size_t)(k0 + r) * D; }, tid);
-  fill_tile<D, kBM>(c.sm + SM::v, nk, [&](int r) { return Vb + (size_t)(k0 + r) * D; }, tid);
+  fill_tile<D, kBM, kKeysThreads>(c.sm + SM::k, nk, [&](int r) { return Kb + (size_t)(k0 + r) * D; }, tid);
+  fill_tile<D, kBM, kKeysThreads>(c.sm + SM::v, nk, [&](int r) { return Vb + (size_t)(k0 + r) * D; }, tid);
   bool started = false;
-  const int u = k0 + tid;
-  TileRegs<D, kBN> qreg, oreg;
+  const int u = k0 + row;
+  TileRegs<D, kBN, kKeysThreads> qreg, oreg;
   float Lreg = 0.f, dreg = 0.f;
   auto load_q = [&](int q0) {
     const int nq = min(kBN, bend - q0);
-    tile_ldg<D, kBN>(qreg, nq, [&](int r) { return Qb + (size_t)(q0 + r) * D; }, tid);
-    tile_ldg<D, kBN>(oreg, nq, [&](int r) { return dOb + (size_t)(q0 + r) * D; }, tid);
+    tile_ldg<D, kBN, kKeysThreads>(qreg, nq, [&](int r) { return Qb + (size_t)(q0 + r) * D; }, tid);
+    tile_ldg<D, kBN, kKeysThreads>(oreg, nq, [&](int r) { return dOb + (size_t)(q0 + r) * D; }, tid);
     if (tid < kBN) {
       Lreg = tid < nq ? LSE[(size_t)pq * dm.N + q0 + tid] * kLog2e : 0.f;
       dreg = tid < nq ? delta[(size_t)pq * dm.N + q0 + tid] : 0.f;
@@ -404,16 +440,16 @@ k_local_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict_
   load_q(k0);
   for (int q0 = k0; q0 < bend && c.ok; q0 += kBN) {
     const int nq = min(kBN, bend - q0);
-    tile_sts<D, kBN>(qreg, c.sm + SM::q, tid);
-    tile_sts<D, kBN>(oreg, c.sm + SM::dO, tid);
+    tile_sts<D, kBN, kKeysThreads>(qreg, c.sm + SM::q, tid);
+    tile_sts<D, kBN, kKeysThreads>(oreg, c.sm + SM::dO, tid);
     if (tid < kBN) { Ls[tid] = Lreg; ds[tid] = dreg; }
-    dkdv_step_tc<D>(c, Ls, ds, [&](int col) { return col < nq && tid < nk && u <= q0 + col; }, dm.sigma * kLog2e, started, tid,
+    dkdv_step_tc<D>(c, Ls, ds, [&](int col) { return col < nq && row < nk && u <= q0 + col; }, dm.sigma * kLog2e, started, tid,
                     [&]() { if (q0 + kBN < bend) load_q(q0 + kBN); });
   }
-  if (c.ok) {
-    const size_t row = ((size_t)pq * dm.N + k0 + tid) * D;
-    read_acc_row<D>(c, 2 * kBN, 1.f, dV_orig + row, tid < nk, tid);
-    read_acc_row<D>(c, 2 * kBN + D, dm.sigma, dK_orig + row, tid < nk, tid);
+  if (c.ok) {                                   // warpgroup 0 writes dV, warpgroup 1 writes dK
+    const size_t at = ((size_t)pq * dm.N + k0 + row) * D;
+    if (wg == 0) read_acc_row<D>(c, 2 * kBN, 1.f, dV_orig + at, row < nk, tid);
+    else read_acc_row<D>(c, 2 * kBN + D, dm.sigma, dK_orig + at, row < nk, tid);
   }
   bwd_teardown(c, SM::cols, tid, status);
 }
@@ -426,7 +462,7 @@ constexpr int kRetSplit = 8;
 
 template <int D>
 __device__ __forceinline__ void add_acc_row(const BwdCtx& c, uint32_t col, float f, float* __restrict__ dst, bool write, int tid) {
-  const uint32_t t = c.tbase + ((uint32_t)((tid >> 5) * 32) << 16) + col;
+  const uint32_t t = c.tbase + ((uint32_t)(((tid >> 5) & 3) * 32) << 16) + col;
 #pragma unroll
   for (int d0 = 0; d0 < D; d0 += 32) {
     float v[32];
@@ -440,7 +476,7 @@ __device__ __forceinline__ void add_acc_row(const BwdCtx& c, uint32_t col, float
 }
 
 template <int D>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kKeysThreads)
 k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO, const bf16* __restrict__ Kp,
                   const bf16* __restrict__ Vp, const float* __restrict__ LSE, const float* __restrict__ delta,
                   const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
@@ -450,8 +486,8 @@ k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
   __shared__ uint64_t bar[2];
   __shared__ uint32_t tbase_s;
   __shared__ __align__(16) float Ls[kBN], ds[kBN];
-  __shared__ int32_t tok_s[kBN];
-  const int tid = threadIdx.x;
+  __shared__ int32_t tok_s[2][kBN];
+  const int tid = threadIdx.x, row = tid & 127, wg = tid >> 7;
   const int j = blockIdx.x, pl = blockIdx.y / kRetSplit, sub = blockIdx.y % kRetSplit, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
@@ -468,50 +504,68 @@ k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
   for (int c0 = kbeg; c0 < kvis && c.ok; c0 += kBM) {
     const int nkc = min(kBM, kvis - c0);
     __syncthreads();
-    fill_tile<D, kBM>(c.sm + SM::k, nkc, [&](int r) { return Kb + (size_t)(c0 + r) * D; }, tid);
-    fill_tile<D, kBM>(c.sm + SM::v, nkc, [&](int r) { return Vb + (size_t)(c0 + r) * D; }, tid);
+    fill_tile<D, kBM, kKeysThreads>(c.sm + SM::k, nkc, [&](int r) { return Kb + (size_t)(c0 + r) * D; }, tid);
+    fill_tile<D, kBM, kKeysThreads>(c.sm + SM::v, nkc, [&](int r) { return Vb + (size_t)(c0 + r) * D; }, tid);
     bool started = false;
-    const bool mine = tid < nkc;
-    TileRegs<D, kBN> qreg, oreg;
+    const bool mine = row < nkc;
+    // Pair ids are fetched two tiles ahead (into tok_s), the rows they point at one tile ahead
+    // (into registers), so neither dependent load sits on the critical path of a tile.
+    TileRegs<D, kBN, kKeysThreads> qreg, oreg;
     float Lreg = 0.f, dreg = 0.f;
-    auto load_pairs = [&](int t) {             // gathers the rows of pair tile t (token = pair id / m)
+    int tokreg = 0;
+    auto load_tokens = [&](int t) {            // thread < 64: token of pair (t, thread), 0 beyond the group
+      if (tid < kBN) { const int t0 = g0 + t * kBN; tokreg = (t < ntiles && t0 + tid < g1) ? __ldg(pr + t0 + tid) / dm.m : 0; }
+    };
+    auto load_rows = [&](int t, const int32_t* tok) {       // tok: shared-memory tokens of tile t
       const int t0 = g0 + t * kBN, nq = min(kBN, g1 - t0);
-      tile_ldg<D, kBN>(qreg, nq, [&](int r) { return Qb + (size_t)(__ldg(pr + t0 + r) / dm.m) * D; }, tid);
-      tile_ldg<D, kBN>(oreg, nq, [&](int r) { return dOb + (size_t)(__ldg(pr + t0 + r) / dm.m) * D; }, tid);
+      tile_ldg<D, kBN, kKeysThreads>(qreg, nq, [&](int r) { return Qb + (size_t)tok[r] * D; }, tid);
+      tile_ldg<D, kBN, kKeysThreads>(oreg, nq, [&](int r) { return dOb + (size_t)tok[r] * D; }, tid);
       if (tid < kBN) {
-        const int tok = tid < nq ? __ldg(pr + t0 + tid) / dm.m : 0;
-        Lreg = tid < nq ? LSE[(size_t)pq * dm.N + tok] * kLog2e : 0.f;
-        dreg = tid < nq ? delta[(size_t)pq * dm.N + tok] : 0.f;
+        Lreg = tid < nq ? LSE[(size_t)pq * dm.N + tok[tid]] * kLog2e : 0.f;
+        dreg = tid < nq ? delta[(size_t)pq * dm.N + tok[tid]] : 0.f;
       }
     };
-    load_pairs(sub);
-    for (int t = sub; t < ntiles && c.ok; t += kRetSplit) {
+    __syncthreads();
+    load_tokens(sub);
+    if (tid < kBN) tok_s[0][tid] = tokreg;
+    load_tokens(sub + kRetSplit);
+    __syncthreads();
+    load_rows(sub, tok_s[0]);
+    int buf = 0;
+    for (int t = sub; t < ntiles && c.ok; t += kRetSplit, buf ^= 1) {
       const int t0 = g0 + t * kBN, nq = min(kBN, g1 - t0);
-      tile_sts<D, kBN>(qreg, c.sm + SM::q, tid);
-      tile_sts<D, kBN>(oreg, c.sm + SM::dO, tid);
-      if (tid < kBN) { Ls[tid] = Lreg; ds[tid] = dreg; }
+      tile_sts<D, kBN, kKeysThreads>(qreg, c.sm + SM::q, tid);
+      tile_sts<D, kBN, kKeysThreads>(oreg, c.sm + SM::dO, tid);
+      if (tid < kBN) { Ls[tid] = Lreg; ds[tid] = dreg; tok_s[buf ^ 1][tid] = tokreg; }     // tokens of the next tile
       dkdv_step_tc<D>(c, Ls, ds, [&](int col) { return col < nq && mine; }, dm.sigma * kLog2e, started, tid,
-                      [&]() { if (t + kRetSplit < ntiles) load_pairs(t + kRetSplit); });
+                      [&]() {                  // runs after the step's first barrier: tok_s[buf ^ 1] is visible
+                        if (t + kRetSplit < ntiles) load_rows(t + kRetSplit, tok_s[buf ^ 1]);
+                        load_tokens(t + 2 * kRetSplit);
+                      });
     }
-    if (c.ok && started) {
-      const size_t row = ((size_t)pq * dm.N + c0 + tid) * D;
-      add_acc_row<D>(c, 2 * kBN, 1.f, dV_perm + row, tid < nkc, tid);
-      add_acc_row<D>(c, 2 * kBN + D, dm.sigma, dK_perm + row, tid < nkc, tid);
+    if (c.ok && started) {                      // warpgroup 0 adds dV, warpgroup 1 adds dK
+      const size_t at = ((size_t)pq * dm.N + c0 + row) * D;
+      if (wg == 0) add_acc_row<D>(c, 2 * kBN, 1.f, dV_perm + at, row < nkc, tid);
+      else add_acc_row<D>(c, 2 * kBN + D, dm.sigma, dK_perm + at, row < nkc, tid);
     }
     tc::fence_before_sync();
   }
+#ifdef MUSE_PHASE_CLOCKS
+  if (tid == 0 && c.pc[5] >= 8 && atomicCAS(status + 40, 0, 1) == 0)
+    for (int k = 0; k < 7; ++k) status[41 + k] = (int)c.pc[k];
+#endif
   bwd_teardown(c, SM::cols, tid, status);
 }
 
 // ---- launchers ------------------------------------------------------------------------------------
-#define MUSE_TC_LAUNCH(KERNEL, SMEM, GRID, ...)                                                                   \
+#define MUSE_TC_LAUNCH(KERNEL, SMEM, NT, GRID, ...)                                                                  \
   do {                                                                                                            \
     if (d.D == 128) {                                                                                             \
       MUSE_CUDA_OK(cudaFuncSetAttribute(KERNEL<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM<128>::total)); \
-      KERNEL<128><<<GRID, 128, SMEM<128>::total, st>>>(__VA_ARGS__);                                              \
+      KERNEL<128><<<GRID, NT, SMEM<128>::total, st>>>(__VA_ARGS__);                                              \
     } else {                                                                                                      \
       MUSE_CUDA_OK(cudaFuncSetAttribute(KERNEL<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM<64>::total));   \
-      KERNEL<64><<<GRID, 128, SMEM<64>::total, st>>>(__VA_ARGS__);                                                \
+      KERNEL<64><<<GRID, NT, SMEM<64>::total, st>>>(__VA_ARGS__);                                                 \
     }                                                                                                             \
     MUSE_LAUNCH_OK();                                                                                             \
   } while (0)
@@ -521,10 +575,10 @@ int local_bwd_tc(const Dims& d, const void* Q, const void* K, const void* V, con
   const int pq = d.B * d.Hq;
   dim3 grid(d.S * cdiv(d.Bs, kBM), pq);
   prof_mark("k_local_bwd_dkdv_tc", st);
-  MUSE_TC_LAUNCH(k_local_bwd_dkdv_tc, KeysSmem, grid, d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, (const bf16*)dO, LSE,
+  MUSE_TC_LAUNCH(k_local_bwd_dkdv_tc, KeysSmem, kKeysThreads, grid, d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, (const bf16*)dO, LSE,
                  delta, dK_orig, dV_orig, status);
   prof_mark("k_local_bwd_dq_tc", st);
-  MUSE_TC_LAUNCH(k_local_bwd_dq_tc, RowsSmem, grid, d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, (const bf16*)dO, LSE,
+  MUSE_TC_LAUNCH(k_local_bwd_dq_tc, RowsSmem, 128, grid, d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, (const bf16*)dO, LSE,
                  delta, dQacc, status);
   return MUSE_OK;
 }
@@ -534,10 +588,10 @@ int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, con
                float* dK_perm, float* dV_perm, int* status, cudaStream_t st) {
   const int pq = d.B * d.Hq;
   prof_mark("k_ret_bwd_dkdv_tc", st);
-  MUSE_TC_LAUNCH(k_ret_bwd_dkdv_tc, KeysSmem, dim3(d.Ck, d.SB * kRetSplit, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
+  MUSE_TC_LAUNCH(k_ret_bwd_dkdv_tc, KeysSmem, kKeysThreads, dim3(d.Ck, d.SB * kRetSplit, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
                  (const bf16*)Vp, LSE, delta, off_k, goff, pairs, dK_perm, dV_perm, status);
   prof_mark("k_ret_bwd_dq_tc", st);
-  MUSE_TC_LAUNCH(k_ret_bwd_dq_tc, RowsSmem, dim3(d.Ck, d.SB * kRetSplitRows, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
+  MUSE_TC_LAUNCH(k_ret_bwd_dq_tc, RowsSmem, 128, dim3(d.Ck, d.SB * kRetSplitRows, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
                  (const bf16*)Vp, LSE, delta, off_k, goff, pairs, (bf16*)dq_part, status);
   return MUSE_OK;
 }

@@ -111,6 +111,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
   for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// 2^x on the special-function unit (about 2 ulp; subnormal results flush to zero)
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 // ---- swizzled shared-memory tiles ------------------------------------------------------------------------
 // Byte offset of the 16-byte chunk `c` (0..7) of row `r` inside a [rows][128 B] tile with the
 // 128-byte swizzle (tile base 1024-byte aligned).
