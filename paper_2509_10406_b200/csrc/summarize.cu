@@ -3,7 +3,13 @@
 // and Causal Accumulation", Eq. 3-5; Algorithm 1 "Causal accumulation along spatial axis").
 #include "common.cuh"
 
+#include <cstdlib>
+
 namespace muse {
+
+bool summarize_tc_supported(const Dims& d, int dtype);
+int summarize_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const float* qbar, const SummPtrs& sp,
+                 int* status, cudaStream_t stream);
 
 SummLayout summ_layout(const Dims& d, int dtype) {
   const size_t es = dtype == MUSE_F32 ? 4 : 2;
@@ -180,6 +186,11 @@ static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const i
   k_gather_rows<T><<<gg, 256, 0, st>>>(V, perm_k, d.N, D, Vp);
   MUSE_LAUNCH_OK();
   if (d.SB == 0) return MUSE_OK;
+  if (summarize_tc_supported(d, dtype) && getenv("MUSE_SUMM_FWD_SIMT") == nullptr) {
+    int32_t* status = (int32_t*)ws + sort_ws_elems(d.N, d.Ck * d.S) * (size_t)pk;      // 64 words after the sort scratch
+    MUSE_CUDA_OK(cudaMemsetAsync(status, 0, 64 * sizeof(int32_t), st));
+    return summarize_tc(d, Kp, Vp, off_k, qbar, summ_ptrs(L, base), status, st);
+  }
   const size_t smem = (size_t)(kSumI * (D + 4) + kSumKC * (2 * D + 4) + kSumI * (kSumKC + 1)) * sizeof(float);
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid(d.Ck, cdiv(d.Cq, kSumI), d.B * d.Hq);
@@ -191,7 +202,7 @@ static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const i
 
 size_t summarize_ws_bytes(const Dims& d) {
   Arena ar(nullptr);
-  ar.take<int32_t>((size_t)d.B * d.Hkv * sort_ws_elems(d.N, d.Ck * d.S));
+  ar.take<int32_t>((size_t)d.B * d.Hkv * sort_ws_elems(d.N, d.Ck * d.S) + 64);
   return ar.used;
 }
 

@@ -1,0 +1,227 @@
+// Accumulated tilted summaries on the tensor cores (bf16 mode, D = 128): Eq. 3-5 and the
+// exclusive causal accumulation of Algorithm 1 in one online-softmax walk over the buckets of a
+// key cluster.  One CTA = (key cluster j, 128 query clusters, head), 256 threads: thread
+// (row i, warpgroup w) keeps the running max / mass of centroid i and 128 fp32 accumulators —
+// the kappa half (w = 0) or the nu half (w = 1).
+//   L   = sigma qbar K^T        tcgen05, qbar as bf16 hi + lo, keys TMA-loaded 64 at a time
+//   w_u = exp(l_u - running max)  per thread, written as a bf16 hi + lo operand pair
+//   U   = W [K | V]             tcgen05 (keys contracted), folded into the accumulators with the
+//                               online-softmax rescale
+// After each bucket the normalised snapshot (mu, beta, kappa hi/lo, nu) of plane = bucket index
+// is staged in shared memory and leaves in coalesced 256-byte rows.
+#include <cuda.h>
+#include "common.cuh"
+#include "tc05.cuh"
+
+namespace muse {
+
+typedef __nv_bfloat16 bf16;
+int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
+
+namespace st {
+constexpr int D = 128, TI = 128, NU = 64, THREADS = 256;
+constexpr int kTile = TI * D * 2, kKeys = NU * D * 2, kW = TI * NU * 2;
+constexpr int oQhi = 0, oQlo = oQhi + kTile, oK = oQlo + kTile, oV = oK + kKeys, oWhi = oV + kKeys, oWlo = oWhi + kW;
+constexpr int total = oWlo + kW + 1024;
+constexpr uint32_t cL = 0, cUk = 64, cUv = 192;
+}  // namespace st
+
+__global__ void __launch_bounds__(st::THREADS, 1)
+k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_constant__ CUtensorMap tm_V,
+               const int32_t* __restrict__ off_k, const float* __restrict__ qbar, SummPtrs sp, int* __restrict__ status) {
+  using namespace st;
+  extern __shared__ __align__(1024) unsigned char sm_raw[];
+  __shared__ uint64_t bar_kv, bar1, bar2;
+  __shared__ uint32_t tbase_s;
+  const int j = blockIdx.x, i0 = blockIdx.y * TI, pq = blockIdx.z;
+  const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
+  const int tid = threadIdx.x, warp = tid >> 5, wg = tid >> 7, row = tid & 127, i = i0 + row;
+  unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
+  const int32_t* off = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
+  if (warp == 0) tc::tmem_alloc(&tbase_s, 512);
+  if (tid == 0) { tc::mbar_init(&bar_kv, 1); tc::mbar_init(&bar1, 1); tc::mbar_init(&bar2, 1); tc::mbar_init_fence(); }
+  // sigma * qbar rows as bf16 hi (warpgroup 0 writes) and lo (warpgroup 1 writes)
+  {
+    const float* src = qbar + ((size_t)pq * dm.Cq + (i < dm.Cq ? i : 0)) * D;
+#pragma unroll
+    for (int ck = 0; ck < D / 8; ++ck) {
+      const float4 f0 = i < dm.Cq ? ld4(src + ck * 8) : make_float4(0.f, 0.f, 0.f, 0.f);
+      const float4 f1 = i < dm.Cq ? ld4(src + ck * 8 + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+      const float x[8] = {f0.x * dm.sigma, f0.y * dm.sigma, f0.z * dm.sigma, f0.w * dm.sigma,
+                          f1.x * dm.sigma, f1.y * dm.sigma, f1.z * dm.sigma, f1.w * dm.sigma};
+      uint32_t w[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        __nv_bfloat162 hh = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]);
+        __nv_bfloat162 ll = __floats2bfloat162_rn(x[2 * e] - __low2float(hh), x[2 * e + 1] - __high2float(hh));
+        w[e] = wg == 0 ? *reinterpret_cast<uint32_t*>(&hh) : *reinterpret_cast<uint32_t*>(&ll);
+      }
+      *reinterpret_cast<uint4*>(sm + (wg == 0 ? oQhi : oQlo) + (ck >> 3) * TI * 128 + tc::sw128_off(row, ck & 7)) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+  }
+  tc::fence_async_smem();
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tbase = tbase_s, tlane = tbase + ((uint32_t)((warp & 3) * 32) << 16);
+  const uint32_t aQhi = tc::smem_u32(sm + oQhi), aQlo = tc::smem_u32(sm + oQlo), aK = tc::smem_u32(sm + oK),
+                 aV = tc::smem_u32(sm + oV), aWhi = tc::smem_u32(sm + oWhi), aWlo = tc::smem_u32(sm + oWlo);
+  uint32_t ph_kv = 0, ph1 = 0, ph2 = 0;
+  bool ok = true;
+  float acc[D];
+#pragma unroll
+  for (int d = 0; d < D; ++d) acc[d] = 0.f;
+  float M = -INFINITY, s = 0.f, T = 0.f;           // running max, mass and sum of w * logit (all relative to M)
+
+  for (int pl = 0; pl < dm.SB && ok; ++pl) {
+    const int p0 = off[pl], p1 = off[pl + 1];
+    for (int c0 = p0; c0 < p1 && ok; c0 += NU) {
+      const int nk = min(NU, p1 - c0);
+      __syncthreads();
+      if (tid == 0) {
+        tc::mbar_expect_tx(&bar_kv, 2 * kKeys);
+        const int r = (int)((size_t)pk * dm.N + c0);
+        tc::tma_load_2d(sm + oK, &tm_K, 0, r, &bar_kv); tc::tma_load_2d(sm + oK + NU * 128, &tm_K, 64, r, &bar_kv);
+        tc::tma_load_2d(sm + oV, &tm_V, 0, r, &bar_kv); tc::tma_load_2d(sm + oV + NU * 128, &tm_V, 64, r, &bar_kv);
+        if (!tc::mbar_wait(&bar_kv, ph_kv)) ok = false;
+        tc::fence_after_sync();
+        const uint32_t idesc = tc::idesc_bf16(TI, NU, 0, 0);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks)
+          tc::mma_bf16_ss(tbase + cL, tc::smem_desc_sw128(aQhi + (ks / 4) * TI * 128 + (ks % 4) * 32, 16, 1024),
+                          tc::smem_desc_sw128(aK + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks)
+          tc::mma_bf16_ss(tbase + cL, tc::smem_desc_sw128(aQlo + (ks / 4) * TI * 128 + (ks % 4) * 32, 16, 1024),
+                          tc::smem_desc_sw128(aK + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, 1);
+        tc::mma_commit(&bar1);
+      }
+      ph_kv ^= 1;
+      __syncwarp();
+      if (!tc::mbar_wait(&bar1, ph1)) ok = false;
+      ph1 ^= 1;
+      tc::fence_after_sync();
+      // two sweeps over the 64 logits in TMEM (max, then weights) keep the register footprint small
+      float cm = -INFINITY;
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        float v[32];
+        tc::tmem_ld32(tlane + cL + 32 * hh, v);
+#pragma unroll
+        for (int u = 0; u < 32; ++u) if (32 * hh + u < nk) cm = fmaxf(cm, v[u]);
+      }
+      const float Mn = fmaxf(M, cm);
+      const float sc = __expf(M - Mn);                 // 0 on the first keys (M = -inf)
+      float ws = 0.f, wl = 0.f;
+#pragma unroll
+      for (int hh = 0; hh < 2; ++hh) {
+        float v[32];
+        tc::tmem_ld32(tlane + cL + 32 * hh, v);
+        uint32_t pk_[16];
+#pragma unroll
+        for (int u = 0; u < 32; u += 2) {
+          const bool in0 = 32 * hh + u < nk, in1 = 32 * hh + u + 1 < nk;
+          const float w0 = in0 ? __expf(v[u] - Mn) : 0.f, w1 = in1 ? __expf(v[u + 1] - Mn) : 0.f;
+          ws += w0 + w1;
+          wl += (in0 ? w0 * v[u] : 0.f) + (in1 ? w1 * v[u + 1] : 0.f);
+          __nv_bfloat162 hb = __floats2bfloat162_rn(w0, w1);
+          __nv_bfloat162 lb = __floats2bfloat162_rn(w0 - __low2float(hb), w1 - __high2float(hb));
+          pk_[u >> 1] = wg == 0 ? *reinterpret_cast<uint32_t*>(&hb) : *reinterpret_cast<uint32_t*>(&lb);
+        }
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch)
+          *reinterpret_cast<uint4*>(sm + (wg == 0 ? oWhi : oWlo) + tc::sw128_off(row, 4 * hh + ch)) = make_uint4(pk_[4 * ch], pk_[4 * ch + 1], pk_[4 * ch + 2], pk_[4 * ch + 3]);
+      }
+      s = s * sc + ws; T = T * sc + wl; M = Mn;
+      tc::fence_async_smem();
+      tc::fence_before_sync();
+      __syncthreads();
+      if (tid == 0) {
+        tc::fence_after_sync();
+        const uint32_t idesc = tc::idesc_bf16(TI, D, 0, 1);          // A = W (K-major over keys), B = key rows (MN-major)
+#pragma unroll
+        for (int ks = 0; ks < NU / 16; ++ks) {
+          tc::mma_bf16_ss(tbase + cUk, tc::smem_desc_sw128(aWhi + ks * 32, 16, 1024), tc::smem_desc_sw128(aK + ks * 16 * 128, NU * 128, 1024), idesc, ks > 0);
+          tc::mma_bf16_ss(tbase + cUv, tc::smem_desc_sw128(aWhi + ks * 32, 16, 1024), tc::smem_desc_sw128(aV + ks * 16 * 128, NU * 128, 1024), idesc, ks > 0);
+        }
+#pragma unroll
+        for (int ks = 0; ks < NU / 16; ++ks) {
+          tc::mma_bf16_ss(tbase + cUk, tc::smem_desc_sw128(aWlo + ks * 32, 16, 1024), tc::smem_desc_sw128(aK + ks * 16 * 128, NU * 128, 1024), idesc, 1);
+          tc::mma_bf16_ss(tbase + cUv, tc::smem_desc_sw128(aWlo + ks * 32, 16, 1024), tc::smem_desc_sw128(aV + ks * 16 * 128, NU * 128, 1024), idesc, 1);
+        }
+        tc::mma_commit(&bar2);
+      }
+      __syncwarp();
+      if (!tc::mbar_wait(&bar2, ph2)) ok = false;
+      ph2 ^= 1;
+      tc::fence_after_sync();
+#pragma unroll
+      for (int d0 = 0; d0 < D; d0 += 32) {
+        float v[32];
+        tc::tmem_ld32(tlane + (wg == 0 ? cUk : cUv) + d0, v);
+#pragma unroll
+        for (int e = 0; e < 32; ++e) acc[d0 + e] = fmaf(acc[d0 + e], sc, v[e]);
+      }
+      tc::fence_before_sync();
+    }
+    // ---- snapshot of plane pl: three 128 x 256-byte row tiles (kappa hi, kappa lo, nu) staged in the W region
+    const bool some = s > 0.f;
+    const float inv = some ? 1.f / s : 0.f;
+    const size_t ent_row0 = ((size_t)pq * dm.SB + pl) * dm.Cq;       // entry = (ent_row0 + i) * Ck + j
+    if (wg == 0 && i < dm.Cq) {
+      const float m_ = some ? M + __logf(s) : -INFINITY;
+      const size_t ent = (ent_row0 + i) * dm.Ck + j;
+      sp.mu[ent] = m_;
+      sp.beta[ent] = some ? m_ - T * inv : -INFINITY;
+    }
+    unsigned char* stage = sm + oWhi;                                 // 32 KB = [128 rows][256 B]
+#pragma unroll
+    for (int round = 0; round < 3; ++round) {                         // 0: kappa hi, 1: kappa lo, 2: nu
+      __syncthreads();
+      if ((round < 2 && wg == 0) || (round == 2 && wg == 1)) {
+#pragma unroll
+        for (int ck = 0; ck < D / 8; ++ck) {
+          uint32_t w[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float x0 = acc[ck * 8 + 2 * e] * inv, x1 = acc[ck * 8 + 2 * e + 1] * inv;
+            __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+            if (round == 1) hh = __floats2bfloat162_rn(x0 - __low2float(hh), x1 - __high2float(hh));
+            w[e] = *reinterpret_cast<uint32_t*>(&hh);
+          }
+          *reinterpret_cast<uint4*>(stage + row * 256 + ((ck ^ (row & 15)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      __syncthreads();
+      bf16* dst = (bf16*)(round == 0 ? sp.khi : round == 1 ? sp.klo : sp.nu);
+      for (int e = tid; e < TI * (D / 8); e += THREADS) {
+        const int r = e >> 4, ck = e & 15;
+        if (i0 + r < dm.Cq) {
+          const uint4 val = *reinterpret_cast<const uint4*>(stage + r * 256 + ((ck ^ (r & 15)) << 4));
+          *reinterpret_cast<uint4*>(dst + ((ent_row0 + i0 + r) * dm.Ck + j) * D + ck * 8) = val;
+        }
+      }
+    }
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tbase, 512);
+  if (!ok && tid == 0) atomicExch(status, 7);
+}
+
+bool summarize_tc_supported(const Dims& d, int dtype) { return dtype == MUSE_BF16 && d.D == st::D; }
+
+int summarize_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const float* qbar, const SummPtrs& sp,
+                 int* status, cudaStream_t stream) {
+  CUtensorMap tK, tV;
+  int rc = make_tmap_bf16_rows(&tK, Kp, (uint64_t)d.B * d.Hkv * d.N, st::D, st::NU);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tV, Vp, (uint64_t)d.B * d.Hkv * d.N, st::D, st::NU);
+  if (rc != MUSE_OK) return rc;
+  MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, st::total));
+  prof_mark("k_summarize_tc", stream);
+  k_summarize_tc<<<dim3(d.Ck, cdiv(d.Cq, st::TI), d.B * d.Hq), st::THREADS, st::total, stream>>>(d, tK, tV, off_k, qbar, sp, status);
+  MUSE_LAUNCH_OK();
+  return MUSE_OK;
+}
+
+}  // namespace muse
