@@ -116,6 +116,8 @@ __device__ __forceinline__ void store_row32(unsigned char* tile, int row, int ha
 // ================================================================================================
 // rows-on-M: dQ of 128 rows (Q, dO tiles already in shared memory) against keys [k_lo, k_hi)
 // ================================================================================================
+constexpr int kRowsThreads = 256;       // rows-on-M kernels: two warpgroups share the 64 key columns
+
 template <int D> struct RowsSmem {
   // the G tile reuses the V tile's bytes: V is dead once the S / dP products have completed
   static constexpr int q = 0, dO = q + kBM * D * 2, k = dO + kBM * D * 2, v = k + kBN * D * 2, g = v,
@@ -127,21 +129,21 @@ template <int D, class Limit>
 __device__ __forceinline__ bool dq_rows_tc(BwdCtx& c, const bf16* __restrict__ Kb, const bf16* __restrict__ Vb, int k_lo,
                                            int k_hi, Limit limit, float scale2, float L2, float delta, int tid) {
   typedef RowsSmem<D> SM;
-  const int warp = tid >> 5;
-  const uint32_t t_s = c.tbase + ((uint32_t)(warp * 32) << 16), t_dp = t_s + kBN;
+  const int warp = tid >> 5, wg = tid >> 7, row = tid & 127;       // 256 threads: warpgroup wg owns key columns [32 wg, +32)
+  const uint32_t t_s = c.tbase + ((uint32_t)((warp & 3) * 32) << 16), t_dp = t_s + kBN;
   const uint32_t qa = tc::smem_u32(c.sm + SM::q), da = tc::smem_u32(c.sm + SM::dO), ka = tc::smem_u32(c.sm + SM::k),
                  va = tc::smem_u32(c.sm + SM::v), ga = tc::smem_u32(c.sm + SM::g);
-  const int my_limit = limit(tid);
+  const int my_limit = limit(row);
   bool first = true;
-  TileRegs<D, kBN> kreg, vreg;
+  TileRegs<D, kBN, kRowsThreads> kreg, vreg;
   if (k_lo < k_hi) {
-    tile_ldg<D, kBN>(kreg, min(kBN, k_hi - k_lo), [&](int r) { return Kb + (size_t)(k_lo + r) * D; }, tid);
-    tile_ldg<D, kBN>(vreg, min(kBN, k_hi - k_lo), [&](int r) { return Vb + (size_t)(k_lo + r) * D; }, tid);
+    tile_ldg<D, kBN, kRowsThreads>(kreg, min(kBN, k_hi - k_lo), [&](int r) { return Kb + (size_t)(k_lo + r) * D; }, tid);
+    tile_ldg<D, kBN, kRowsThreads>(vreg, min(kBN, k_hi - k_lo), [&](int r) { return Vb + (size_t)(k_lo + r) * D; }, tid);
   }
   for (int c0 = k_lo; c0 < k_hi && c.ok; c0 += kBN) {
     const int nk = min(kBN, k_hi - c0);
-    tile_sts<D, kBN>(kreg, c.sm + SM::k, tid);
-    tile_sts<D, kBN>(vreg, c.sm + SM::v, tid);
+    tile_sts<D, kBN, kRowsThreads>(kreg, c.sm + SM::k, tid);
+    tile_sts<D, kBN, kRowsThreads>(vreg, c.sm + SM::v, tid);
     tc::fence_async_smem();
     tc::fence_before_sync();
     __syncthreads();
@@ -156,26 +158,24 @@ __device__ __forceinline__ bool dq_rows_tc(BwdCtx& c, const bf16* __restrict__ K
     }
     if (c0 + kBN < k_hi) {                   // next key tile: loads fly while the MMAs and the softmax piece run
       const int cn = c0 + kBN, nn = min(kBN, k_hi - cn);
-      tile_ldg<D, kBN>(kreg, nn, [&](int r) { return Kb + (size_t)(cn + r) * D; }, tid);
-      tile_ldg<D, kBN>(vreg, nn, [&](int r) { return Vb + (size_t)(cn + r) * D; }, tid);
+      tile_ldg<D, kBN, kRowsThreads>(kreg, nn, [&](int r) { return Kb + (size_t)(cn + r) * D; }, tid);
+      tile_ldg<D, kBN, kRowsThreads>(vreg, nn, [&](int r) { return Vb + (size_t)(cn + r) * D; }, tid);
     }
     if (!tc::mbar_wait(&c.bar[0], c.ph0)) { c.ok = false; break; }
     c.ph0 ^= 1;
     tc::fence_after_sync();
     const int vis = min(nk, my_limit - c0 + 1);
-    float g[kBN];
-#pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      float s[32], dp[32];
-      tc::tmem_ld32(t_s + 32 * h, s);
-      tc::tmem_ld32(t_dp + 32 * h, dp);
+    {
+      float s[32], dp[32], g[32];
+      tc::tmem_ld32(t_s + 32 * wg, s);
+      tc::tmem_ld32(t_dp + 32 * wg, dp);
 #pragma unroll
       for (int i = 0; i < 32; ++i) {
-        const float p = (32 * h + i) < vis ? tc::fast_exp2(s[i] * scale2 - L2) : 0.f;
-        g[32 * h + i] = p * (dp[i] - delta);
+        const float e = tc::fast_exp2(s[i] * scale2 - L2);
+        g[i] = ((32 * wg + i) < vis ? e : 0.f) * (dp[i] - delta);
       }
+      store_row32(c.sm + SM::g, row, wg, g);
     }
-    store_row64(c.sm + SM::g, tid, g);
     tc::fence_async_smem();
     tc::fence_before_sync();
     __syncthreads();
@@ -214,14 +214,14 @@ __device__ __forceinline__ void read_acc_row(const BwdCtx& c, uint32_t col, floa
 }
 
 template <int D>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kRowsThreads)
 k_local_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ K, const bf16* __restrict__ V,
                   const bf16* __restrict__ dO, const float* __restrict__ LSE, const float* __restrict__ delta,
                   float* __restrict__ dQacc, int* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar[2];
   __shared__ uint32_t tbase_s;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x, row = tid & 127, wg = tid >> 7;
   BwdCtx c;
   bwd_setup(c, sm_raw, bar, &tbase_s, RowsSmem<D>::cols, tid);
   const int tpb = cdiv(dm.Bs, kBM);
@@ -231,19 +231,19 @@ k_local_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
   const int q0 = bstart + qt * kBM, nq = min(kBM, bend - q0);
   const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
   const bf16* Kb = K + (size_t)pk * dm.N * D; const bf16* Vb = V + (size_t)pk * dm.N * D;
-  fill_tile<D, kBM>(c.sm + RowsSmem<D>::q, nq, [&](int r) { return Qb + (size_t)(q0 + r) * D; }, tid);
-  fill_tile<D, kBM>(c.sm + RowsSmem<D>::dO, nq, [&](int r) { return dOb + (size_t)(q0 + r) * D; }, tid);
-  const size_t t = (size_t)pq * dm.N + q0 + tid;
-  const float L2 = tid < nq ? LSE[t] * kLog2e : 0.f, dl = tid < nq ? delta[t] : 0.f;
+  fill_tile<D, kBM, kRowsThreads>(c.sm + RowsSmem<D>::q, nq, [&](int r) { return Qb + (size_t)(q0 + r) * D; }, tid);
+  fill_tile<D, kBM, kRowsThreads>(c.sm + RowsSmem<D>::dO, nq, [&](int r) { return dOb + (size_t)(q0 + r) * D; }, tid);
+  const size_t t = (size_t)pq * dm.N + q0 + row;
+  const float L2 = row < nq ? LSE[t] * kLog2e : 0.f, dl = row < nq ? delta[t] : 0.f;
   dq_rows_tc<D>(c, Kb, Vb, bstart, q0 + nq, [&](int r) { return q0 + r; }, dm.sigma * kLog2e, L2, dl, tid);
-  if (c.ok) read_acc_row<D>(c, 2 * kBN, dm.sigma, dQacc + t * D, tid < nq, tid);
+  if (c.ok) read_acc_row<D / 2>(c, 2 * kBN + wg * (D / 2), dm.sigma, dQacc + t * D + wg * (D / 2), row < nq, tid);   // each warpgroup half a row
   bwd_teardown(c, RowsSmem<D>::cols, tid, status);
 }
 
 constexpr int kRetSplitRows = 4;      // CTAs sharing the 128-pair tiles of one (cluster, plane) group
 
 template <int D>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kRowsThreads)
 k_ret_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO, const bf16* __restrict__ Kp,
                 const bf16* __restrict__ Vp, const float* __restrict__ LSE, const float* __restrict__ delta,
                 const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
@@ -251,14 +251,14 @@ k_ret_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar[2];
   __shared__ uint32_t tbase_s;
-  __shared__ int32_t pid_s[kBM];
-  const int tid = threadIdx.x;
+  __shared__ int32_t pid_s[2][kBM];
+  const int tid = threadIdx.x, row = tid & 127, wg = tid >> 7;
   const int j = blockIdx.x, pl = blockIdx.y / kRetSplitRows, sub = blockIdx.y % kRetSplitRows, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
   const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)pl * dm.Ck + j;
-  const int g0 = go[0], g1 = go[1];
-  if (g0 + sub * kBM >= g1) return;                   // this split has no pair tile
+  const int g0 = go[0], g1 = go[1], ntiles = (g1 - g0 + kBM - 1) / kBM;
+  if (sub >= ntiles) return;                          // this split has no pair tile
   const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const int k0 = ok[0], k1 = ok[pl + 1];
   BwdCtx c;
@@ -266,24 +266,47 @@ k_ret_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO
   const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
   const bf16* Kb = Kp + (size_t)pk * dm.N * D; const bf16* Vb = Vp + (size_t)pk * dm.N * D;
   const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
-  for (int t0 = g0 + sub * kBM; t0 < g1 && c.ok; t0 += kRetSplitRows * kBM) {
-    const int nq = min(kBM, g1 - t0);
-    __syncthreads();
-    pid_s[tid] = tid < nq ? pr[t0 + tid] : 0;
-    __syncthreads();
-    fill_tile<D, kBM>(c.sm + RowsSmem<D>::q, nq, [&](int r) { return Qb + (size_t)(pid_s[r] / dm.m) * D; }, tid);
-    fill_tile<D, kBM>(c.sm + RowsSmem<D>::dO, nq, [&](int r) { return dOb + (size_t)(pid_s[r] / dm.m) * D; }, tid);
-    const size_t t = (size_t)pq * dm.N + pid_s[tid] / dm.m;
-    const float L2 = tid < nq ? LSE[t] * kLog2e : 0.f, dl = tid < nq ? delta[t] : 0.f;
+  // pair ids two tiles ahead (shared memory), the rows they point at one tile ahead (registers)
+  TileRegs<D, kBM, kRowsThreads> qreg, oreg;
+  float Lreg = 0.f, dreg = 0.f;
+  int pidreg = 0;
+  auto load_pids = [&](int t) {
+    if (tid < kBM) { const int t0 = g0 + t * kBM; pidreg = (t < ntiles && t0 + tid < g1) ? __ldg(pr + t0 + tid) : 0; }
+  };
+  auto load_rows = [&](int t, const int32_t* pid) {
+    const int t0 = g0 + t * kBM, nq = min(kBM, g1 - t0);
+    tile_ldg<D, kBM, kRowsThreads>(qreg, nq, [&](int r) { return Qb + (size_t)(pid[r] / dm.m) * D; }, tid);
+    tile_ldg<D, kBM, kRowsThreads>(oreg, nq, [&](int r) { return dOb + (size_t)(pid[r] / dm.m) * D; }, tid);
+    const size_t tt = (size_t)pq * dm.N + pid[row] / dm.m;
+    Lreg = row < nq ? LSE[tt] * kLog2e : 0.f;
+    dreg = row < nq ? delta[tt] : 0.f;
+  };
+  load_pids(sub);
+  if (tid < kBM) pid_s[0][tid] = pidreg;
+  load_pids(sub + kRetSplitRows);
+  __syncthreads();
+  load_rows(sub, pid_s[0]);
+  int buf = 0;
+  for (int t = sub; t < ntiles && c.ok; t += kRetSplitRows, buf ^= 1) {
+    const int t0 = g0 + t * kBM, nq = min(kBM, g1 - t0);
+    tile_sts<D, kBM, kRowsThreads>(qreg, c.sm + RowsSmem<D>::q, tid);
+    tile_sts<D, kBM, kRowsThreads>(oreg, c.sm + RowsSmem<D>::dO, tid);
+    if (tid < kBM) pid_s[buf ^ 1][tid] = pidreg;                      // pair ids of the next tile
+    const float L2 = Lreg, dl = dreg;
+    const int my_pid = pid_s[buf][row];
+    __syncthreads();                                                  // pid_s[buf ^ 1] visible before the prefetch below
+    if (t + kRetSplitRows < ntiles) load_rows(t + kRetSplitRows, pid_s[buf ^ 1]);
+    load_pids(t + 2 * kRetSplitRows);
     const bool any = dq_rows_tc<D>(c, Kb, Vb, k0, k1, [&](int) { return k1 - 1; }, dm.sigma * kLog2e, L2, dl, tid);
     if (c.ok) {
-      bf16* dst = dq_part + ((size_t)pq * dm.N * dm.m + pid_s[tid]) * D;       // bf16 row per (query, slot)
-      const uint32_t tq = c.tbase + ((uint32_t)((tid >> 5) * 32) << 16) + 2 * kBN;
+      // bf16 row per (query, slot); each warpgroup converts and stores half of it
+      bf16* dst = dq_part + ((size_t)pq * dm.N * dm.m + my_pid) * D + wg * (D / 2);
+      const uint32_t tq = c.tbase + ((uint32_t)(((tid >> 5) & 3) * 32) << 16) + 2 * kBN + wg * (D / 2);
 #pragma unroll
-      for (int d0 = 0; d0 < D; d0 += 32) {
+      for (int d0 = 0; d0 < D / 2; d0 += 32) {
         float v[32];
         if (any) tc::tmem_ld32(tq + d0, v);
-        if (tid < nq) {
+        if (row < nq) {
 #pragma unroll
           for (int i = 0; i < 32; i += 8) {
             uint32_t w[4];
@@ -578,7 +601,7 @@ int local_bwd_tc(const Dims& d, const void* Q, const void* K, const void* V, con
   MUSE_TC_LAUNCH(k_local_bwd_dkdv_tc, KeysSmem, kKeysThreads, grid, d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, (const bf16*)dO, LSE,
                  delta, dK_orig, dV_orig, status);
   prof_mark("k_local_bwd_dq_tc", st);
-  MUSE_TC_LAUNCH(k_local_bwd_dq_tc, RowsSmem, 128, grid, d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, (const bf16*)dO, LSE,
+  MUSE_TC_LAUNCH(k_local_bwd_dq_tc, RowsSmem, kRowsThreads, grid, d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, (const bf16*)dO, LSE,
                  delta, dQacc, status);
   return MUSE_OK;
 }
@@ -591,7 +614,7 @@ int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, con
   MUSE_TC_LAUNCH(k_ret_bwd_dkdv_tc, KeysSmem, kKeysThreads, dim3(d.Ck, d.SB * kRetSplit, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
                  (const bf16*)Vp, LSE, delta, off_k, goff, pairs, dK_perm, dV_perm, status);
   prof_mark("k_ret_bwd_dq_tc", st);
-  MUSE_TC_LAUNCH(k_ret_bwd_dq_tc, RowsSmem, 128, dim3(d.Ck, d.SB * kRetSplitRows, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
+  MUSE_TC_LAUNCH(k_ret_bwd_dq_tc, RowsSmem, kRowsThreads, dim3(d.Ck, d.SB * kRetSplitRows, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
                  (const bf16*)Vp, LSE, delta, off_k, goff, pairs, (bf16*)dq_part, status);
   return MUSE_OK;
 }
