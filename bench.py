@@ -39,25 +39,44 @@ def work_model(w: wl.Workload):
     e = 4 if w.dtype == "f32" else 2
     Bs, SB = N // S, S - 1
     heads, kvh = B * Hq, B * Hkv
-    summ = heads * SB * Cq * Ck * (2 * D + 1) * 4           # accumulated summaries, fp32
     nd = N * D
     ret_keys = m * (N / Ck) * (S - 1) / (2 * S)             # nominal retrieved keys per query
     local = 2 * D * N * Bs                                  # 2 matmuls over the causal half
+    far_tc = w.dtype == "bf16" and D == 128 and Ck % 128 == 0 and Ck <= 1024      # tensor-core far-field path
+    summ = heads * SB * Cq * Ck * ((3 * D * 2 + 8) if far_tc else (2 * D + 1) * 4)  # accumulated summaries
+    grads = heads * SB * Cq * Ck * ((2 * D * 2 + 4) if far_tc else (2 * D + 1) * 4) # their gradients
+    part = heads * N * m * D * (2 if w.dtype == "bf16" else 4)                       # retrieval partials (o or dq)
     M = {
+        # clustering
         "k_assign": ("tensor", 2.0 * N * D * (T + 1) * (Cq * heads + Ck * kvh)),
+        "k_assign_tc": ("tensor", 2.0 * N * D * (T + 1) * (Cq * heads + Ck * kvh)),
         "k_update": ("hbm", T * (heads + kvh) * nd * e),
         "k_gather_rows": ("hbm", 2 * kvh * nd * e * 2),
+        # summaries: bound by the write of the summaries
         "k_summarize": ("hbm", summ + 2 * kvh * nd * e),
+        "k_summarize_tc": ("hbm", summ + 2 * kvh * nd * e),
+        # far field: bound by the read of the summaries
         "k_far_fwd": ("hbm", summ + heads * nd * (e + 4)),
+        "k_far_fwd_tc": ("hbm", summ + heads * nd * (e + 4)),
+        "k_far_bwd": ("hbm", summ + grads + heads * nd * (2 * e + 8)),
+        "k_far_bwd_tc": ("hbm", summ + grads + heads * nd * (2 * e + 8)),
+        "k_summ_bwd": ("hbm", grads + 2 * kvh * nd * e + 4 * heads * nd * 4),
+        "k_summ_bwd_tc": ("hbm", grads + 2 * kvh * nd * e + 4 * heads * nd * 4),
+        # exact attention: tensor bound
         "k_local_fwd": ("tensor", heads * float(local)),
+        "k_local_fwd_tc": ("tensor", heads * float(local)),
+        "k_local_bwd_dkdv": ("tensor", heads * 2.0 * local),      # S, dP, dV, dK
+        "k_local_bwd_dkdv_tc": ("tensor", heads * 2.0 * local),
+        "k_local_bwd_dq": ("tensor", heads * 1.5 * local),        # S, dP, dQ
+        "k_local_bwd_dq_tc": ("tensor", heads * 1.5 * local),
         "k_ret_fwd": ("tensor", heads * 4.0 * D * N * ret_keys),
-        "k_merge": ("hbm", heads * (nd * (8 + e) + N * m * (D + 1) * 4)),
-        "k_local_bwd_dkdv": ("tensor", heads * 2.0 * local),   # S, dP, dV, dK
-        "k_local_bwd_dq": ("tensor", heads * 1.5 * local),     # S, dP, dQ
+        "k_ret_fwd_tc": ("tensor", heads * 4.0 * D * N * ret_keys),
         "k_ret_bwd": ("tensor", heads * 10.0 * D * N * ret_keys),
-        "k_far_bwd": ("hbm", 2 * summ + heads * nd * (2 * e + 8)),
-        "k_summ_bwd": ("hbm", summ + 2 * kvh * nd * e + 4 * heads * nd * 4),
-        "k_final_dq": ("hbm", heads * (nd * (4 + e) + N * m * D * 4)),
+        "k_ret_bwd_dkdv_tc": ("tensor", heads * 8.0 * D * N * ret_keys),
+        "k_ret_bwd_dq_tc": ("tensor", heads * 6.0 * D * N * ret_keys),
+        # merges and assembly
+        "k_merge": ("hbm", heads * nd * (8 + e) + part + heads * N * m * 4),
+        "k_final_dq": ("hbm", heads * nd * (4 + e) + part),
         "k_final_dkv": ("hbm", heads * 4 * nd * 4 + kvh * 2 * nd * e),
     }
     return M

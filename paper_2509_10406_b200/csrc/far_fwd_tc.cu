@@ -201,9 +201,20 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
             uint32_t kmx = 0u, kmn = 0xffffffffu;
 #pragma unroll
             for (int k = 0; k < 32; ++k) { kmx = max(kmx, key[k]); kmn = min(kmn, key[k] >= kFinite ? key[k] : 0xffffffffu); }
+            const uint32_t lane_max = kmx;
             kmx = __reduce_max_sync(0xffffffffu, kmx);
             kmn = __reduce_min_sync(0xffffffffu, kmn);
-            const int shared = __clz((int)(kmx ^ kmn));            // 32 if all finite keys are equal
+            if (m <= 32) {
+              // the m-th largest of the 32 lane maxima bounds the m-th largest score from below:
+              // a cheap one-value-per-lane bisection that shortens the search interval
+              uint32_t lb = 0;
+              for (int bit = 31; bit >= 0; --bit) {
+                const uint32_t cand = lb | (1u << bit);
+                if (__popc(__ballot_sync(0xffffffffu, lane_max >= cand)) >= m) lb = cand;
+              }
+              kmn = max(kmn, lb);
+            }
+            const int shared = __clz((int)(kmx ^ kmn));            // 32 if the interval is a single key
             T = shared >= 32 ? kmx : (kmx & ~(0xffffffffu >> shared));
             for (int bit = 31 - shared; bit >= 0; --bit) {
               const uint32_t cand = T | (1u << bit);
