@@ -210,6 +210,13 @@ def workload_config(w, gain):
             "parallelism": "replicas"}
 
 
+# DRAM bytes per (batch, head) problem from the ncu capture of the headline workload cut to one
+# head (dram__bytes_read.sum + dram__bytes_write.sum; the capture's command and figures are in
+# profiles/top_kernels_headline_one_head.md).  Traffic grows in proportion to the problem count.
+NCU_TRAFFIC_PER_HEAD = {"k_summarize_tc": 1.446e9, "k_local_fwd_tc": 0.0535e9, "k_far_fwd_tc": 2.145e9,
+                        "k_ret_bwd_dkdv_tc": 0.0494e9, "k_far_bwd_tc": 2.374e9, "k_summ_bwd_tc": 1.165e9}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -220,6 +227,10 @@ def main():
     ap.add_argument("--gain", type=float, default=1.0, help="multiplier on Q (1 = literal workload)")
     ap.add_argument("--m", type=int, default=None, help="override retrieved clusters per query")
     ap.add_argument("--heads", type=int, default=None, help="override head count (smaller captures)")
+    ap.add_argument("--head-groups", type=int, default=0,
+                    help="run the KV-head groups in this many sequential stages over one set of buffers "
+                         "(0 = as few as keep the summaries under 64 GB)")
+    ap.add_argument("--forward-only", action="store_true", help="time cluster + summarize + forward only")
     ap.add_argument("--ref-rows", type=int, default=128, help="sampled queries for the oracle timing")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
@@ -255,17 +266,36 @@ def main():
     hQ, hK, hV, hdO = pin(Qh), pin(Kh), pin(Vh), pin(dOh)
     Q, K, V, dO = (x.cuda(non_blocking=True) for x in (hQ, hK, hV, hdO))
     init_q, init_k = torch.from_numpy(iq).cuda(), torch.from_numpy(ik).cuda()
-    p = mb.make_params(B=w.B, Hq=w.Hq, Hkv=w.Hkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=w.m, n_blocks=w.S,
+    # Head staging: every KV-head group is an independent problem, so a layer whose summaries do
+    # not fit the device at once runs its groups one after another over one set of buffers.
+    groups = args.head_groups
+    if groups <= 0:
+        full = mb.make_params(B=w.B, Hq=w.Hq, Hkv=w.Hkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=w.m, n_blocks=w.S,
+                              dtype=w.dtype, kmeans_iters=w.T)
+        need = mb.muse_workspace_bytes(full)[4]
+        groups = 1
+        while need / groups > 64e9 and groups < w.Hkv:
+            groups *= 2
+    if groups > 1 and (w.B != 1 or w.Hkv % groups):
+        raise SystemExit("head staging needs B == 1 and a group count that divides the KV heads")
+    hq, hkv = w.Hq // groups, w.Hkv // groups
+    p = mb.make_params(B=w.B, Hq=hq, Hkv=hkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=w.m, n_blocks=w.S,
                        dtype=w.dtype, kmeans_iters=w.T)
-    buf = mb.MuseBuffers(p, backward=True)
+    buf = mb.MuseBuffers(p, backward=not args.forward_only)
+    O_all = torch.empty_like(Q)
+    dQ_all, dK_all, dV_all = (None, None, None) if args.forward_only else (torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V))
 
     def step():
-        mb.muse_cluster(p, Q, K, init_q, init_k, buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, buf.ws)
-        mb.muse_summarize(p, K, V, buf.assign_k, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
-        mb.muse_attn_fwd(p, Q, K, V, buf.assign_q, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, None, buf.O,
-                         buf.LSE, buf.sel, buf.ws)
-        mb.muse_attn_bwd(p, Q, K, V, buf.O, buf.LSE, dO, buf.assign_q, buf.qbar, buf.off_k, buf.perm_k,
-                         buf.summaries, buf.sel, buf.dQ, buf.dK, buf.dV, buf.ws)
+        for g in range(groups):
+            qs, ks = slice(g * hq, (g + 1) * hq), slice(g * hkv, (g + 1) * hkv)
+            Qg, Kg, Vg = Q[:, qs], K[:, ks], V[:, ks]
+            mb.muse_cluster(p, Qg, Kg, init_q[:, qs], init_k[:, ks], buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, buf.ws)
+            mb.muse_summarize(p, Kg, Vg, buf.assign_k, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
+            mb.muse_attn_fwd(p, Qg, Kg, Vg, buf.assign_q, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, None,
+                             O_all[:, qs], buf.LSE, buf.sel, buf.ws)
+            if not args.forward_only:
+                mb.muse_attn_bwd(p, Qg, Kg, Vg, O_all[:, qs], buf.LSE, dO[:, qs], buf.assign_q, buf.qbar, buf.off_k,
+                                 buf.perm_k, buf.summaries, buf.sel, dQ_all[:, qs], dK_all[:, ks], dV_all[:, ks], buf.ws)
 
     def barrier():
         if world > 1:
@@ -301,15 +331,18 @@ def main():
     # end to end: host buffers in, host buffers out, through the same public calls
     e2e = None
     if not args.no_e2e:
-        hO, hdQ = torch.empty_like(hQ), torch.empty_like(hQ)
-        hdK, hdV = torch.empty_like(hK), torch.empty_like(hK)
+        hO = torch.empty_like(hQ)
+        outs = [(hO, O_all)]
+        if not args.forward_only:
+            hdQ, hdK, hdV = torch.empty_like(hQ), torch.empty_like(hK), torch.empty_like(hK)
+            outs += [(hdQ, dQ_all), (hdK, dK_all), (hdV, dV_all)]
 
         def e2e_step():
             Q.copy_(hQ, non_blocking=True); K.copy_(hK, non_blocking=True)
             V.copy_(hV, non_blocking=True); dO.copy_(hdO, non_blocking=True)
             step()
-            hO.copy_(buf.O, non_blocking=True); hdQ.copy_(buf.dQ, non_blocking=True)
-            hdK.copy_(buf.dK, non_blocking=True); hdV.copy_(buf.dV, non_blocking=True)
+            for h, d in outs:
+                h.copy_(d, non_blocking=True)
         e2e_step()
         barrier()
         ev0.record()
@@ -324,7 +357,7 @@ def main():
             ems = float(t.item())
         nb = lambda *ts: int(sum(x.numel() * x.element_size() for x in ts))
         e2e = {"value": world * tokens / (ems * 1e-3), "unit": UNIT, "ms_per_step": ems,
-               "h2d_bytes_per_step": nb(hQ, hK, hV, hdO), "d2h_bytes_per_step": nb(hO, hdQ, hdK, hdV)}
+               "h2d_bytes_per_step": nb(hQ, hK, hV, hdO), "d2h_bytes_per_step": nb(*[h for h, _ in outs])}
 
     if rank != 0:
         if world > 1:
@@ -347,7 +380,10 @@ def main():
             ach, peak, unit = work / sec / 1e12, pk["tensor_sustained"], "TFLOP/s"
         else:
             ach, peak, unit = work / sec / 1e9, pk["hbm"], "GB/s"
-        roof.update(bound=bound, achieved=ach, peak=peak, unit=unit, frac=ach / peak, traffic=None,
+        traffic = None
+        if w.name == "headline" and args.m is None and top in NCU_TRAFFIC_PER_HEAD:
+            traffic = NCU_TRAFFIC_PER_HEAD[top] * w.B * w.Hq    # one launch per step covers all heads
+        roof.update(bound=bound, achieved=ach, peak=peak, unit=unit, frac=ach / peak, traffic=traffic,
                     peak_source=pk["source"] + (" (sustained bf16)" if bound == "tensor" else " (copy)"),
                     algorithmic_work_per_step=work, kernel_ms_per_step=kernels[top]["ms_per_step"])
     for k, v in kernels.items():
@@ -392,7 +428,10 @@ def main():
 
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype,
-            "data": "synthetic", "config": workload_config(w, args.gain), "clocks": clocks, "e2e": e2e,
+            "data": "synthetic",
+            "config": dict(workload_config(w, args.gain), head_stages=groups,
+                           passes="cluster+summarize+forward" if args.forward_only else "cluster+summarize+forward+backward"),
+            "clocks": clocks, "e2e": e2e,
             "gpu_launches": launches, "roofline": roof, "cpu_baseline": cpu, "kernels": kernels, "context": context}
     print(json.dumps(line))
     if world > 1:
