@@ -30,7 +30,10 @@ summaries; m = C_k, singleton key clusters or singleton query clusters give
 dense causal softmax attention (textbook formula written separately in the
 test); key-translation invariance; weights sum to one and are causal;
 error bilinear in the residuals; backward vs central finite differences and,
-for m = C_k, vs the closed-form dense-attention gradient.
+for m = C_k, vs the closed-form dense-attention gradient.  Dipole: the Jacobian
+of the far field at zero residual equals the dense-attention Jacobian (a
+cross-covariance written separately in the test), the error falls from first
+to second order in the residual, causality and key-translation invariance.
 """
 from __future__ import annotations
 
@@ -40,6 +43,7 @@ __all__ = [
     "lloyd", "assign_nearest", "assignment_gaps", "strided_init", "feistel_permute",
     "block_summaries", "accumulate", "accumulated_summaries",
     "select_clusters", "forward", "backward", "layer_forward", "layer_backward",
+    "untilted_covariances", "merged_dipole",
 ]
 
 _M64 = (1 << 64) - 1
@@ -204,6 +208,52 @@ def accumulated_summaries(K, V, a_k, qbar, sigma, S, Ck, causal=True):
 
 
 # --------------------------------------------------------------------------------------------
+# Dipole correction (Appendix "Error Analysis", paragraphs "Dipole Correction" and "Untilted
+# (Partially Specialized) Covariances")
+# --------------------------------------------------------------------------------------------
+
+def untilted_covariances(K, V, a_k, S, Ck, causal=True):
+    """Shared, untilted within-cluster cross-covariance of values and keys, one per key cluster
+    and spatial block: over M_jb = {u : a_k[u] = j, block(u) < b} with uniform weights,
+    Cov_0jb(v,k) = mean(v k^T) - mean(v) mean(k)^T  (rows = value dims, columns = key dims).
+    Empty sets give zero.  Shape [S, Ck, Dv, D]."""
+    K = np.asarray(K, np.float64); V = np.asarray(V, np.float64)
+    N, D = K.shape; Dv = V.shape[1]
+    if not causal:
+        S = 1
+    Bs = N // S
+    blk = np.arange(N) // Bs
+    cov = np.zeros((S, Ck, Dv, D))
+    for b in range(S):
+        vis = (blk < b) if causal else np.ones(N, bool)
+        for j in range(Ck):
+            mem = np.nonzero(vis & (a_k == j))[0]
+            if mem.size == 0:
+                continue
+            k, v = K[mem], V[mem]
+            cov[b, j] = v.T @ k / mem.size - np.outer(v.mean(0), k.mean(0))
+    return cov
+
+
+def merged_dipole(muh, cov):
+    """Pre-merged dipole matrix per query cluster and block: Cbar_ib = sum_j p_ib(j) Cov_0jb
+    with the centroid attention weights p_ib(j) = softmax_j muh_ijb over the non-empty key
+    clusters.  muh [S,Cq,Ck], cov [S,Ck,Dv,D] -> [S,Cq,Dv,D]; zero where no cluster is visible."""
+    S, Cq, Ck = muh.shape
+    cbar = np.zeros((S, Cq) + cov.shape[2:])
+    for b in range(S):
+        for i in range(Cq):
+            fin = np.isfinite(muh[b, i])
+            if not fin.any():
+                continue
+            mx = muh[b, i][fin].max()
+            p = np.where(fin, np.exp(np.where(fin, muh[b, i], mx) - mx), 0.0)
+            p /= p.sum()
+            cbar[b, i] = np.tensordot(p, cov[b], axes=(0, 0))
+    return cbar
+
+
+# --------------------------------------------------------------------------------------------
 # Per-query attention (Section "Two-Level Retrieval", Eq. 6; "Exact Retrieval and Local
 # Attention"; "Output merging")
 # --------------------------------------------------------------------------------------------
@@ -242,7 +292,7 @@ def _softmax_part(logits, values):
 
 
 def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs, m, causal,
-             sel_rows, sel_mode):
+             sel_rows, sel_mode, cbar_ib=None):
     """All quantities of Algorithm 1's per-query loop for the queries `rows`, which share the
     query cluster (centroid qbar_i) and the spatial block b."""
     N = K.shape[0]
@@ -269,6 +319,9 @@ def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs
     # 1. far field: approximate attention over the clusters that were not retrieved
     far_logit = np.where(nonempty[None, :] & ~selmask, score, -np.inf)
     o_far, lse_far = _softmax_part(far_logit, nuh_ib)
+    if cbar_ib is not None:
+        # dipole: the linear value term, merged over clusters; the mass (lse_far) is unchanged
+        o_far = o_far + np.where(np.isfinite(lse_far)[:, None], qres @ cbar_ib.T, 0.0)
     # 3. exact attention over the retrieved clusters' visible keys (full query)
     u = np.arange(N)
     vis = (u // Bs < b) if causal else np.ones(N, bool)
@@ -305,10 +358,14 @@ def _segments(a_q, N, S, causal, rows):
 
 
 def forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, sel_mode=0,
-            summ=None, rows=None):
+            summ=None, rows=None, dipole=0):
     """MuSe attention for one head.  Returns a dict with O [N,Dv], LSE [N], sel [N,m] and the
     three component (o, lse) pairs.  `sel` forces the retrieved clusters (teacher forcing);
-    `rows` restricts the computation to some queries (others are left zero / -inf / -1)."""
+    `rows` restricts the computation to some queries (others are left zero / -inf / -1).
+    `dipole=1` adds the untilted pre-merged dipole correction to the far field; the paper
+    defines it without retrieval, so it requires m = 0."""
+    if dipole and m != 0:
+        raise ValueError("the dipole correction is defined for m = 0 (no retrieval)")
     Q = np.asarray(Q, np.float64); K = np.asarray(K, np.float64); V = np.asarray(V, np.float64)
     qbar = np.asarray(qbar, np.float64)
     N, D = Q.shape; Dv = V.shape[1]
@@ -318,6 +375,7 @@ def forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, 
     if summ is None:
         summ = accumulated_summaries(K, V, a_k, qbar, sigma, S, Ck, causal)
     muh, kah, nuh = summ
+    cbar = merged_dipole(muh, untilted_covariances(K, V, a_k, S, Ck, causal)) if dipole else None
     out = dict(O=np.zeros((N, Dv)), LSE=np.full(N, -np.inf), sel=np.full((N, m), -1, np.int32),
                sel_gap=np.full(N, np.inf))
     for name in ("o_far", "o_ret", "o_loc"):
@@ -327,12 +385,14 @@ def forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, 
     for b, i, r in _segments(a_q, N, S, causal, rows):
         seg = _segment(Q, K, V, a_k, qbar[i], muh[b, i], kah[b, i], nuh[b, i], r, b,
                        sigma=sigma, Bs=Bs, m=m, causal=causal,
-                       sel_rows=None if sel is None else sel[r], sel_mode=sel_mode)
+                       sel_rows=None if sel is None else sel[r], sel_mode=sel_mode,
+                       cbar_ib=None if cbar is None else cbar[b, i])
         out["O"][r], out["LSE"][r], out["sel"][r] = seg["O"], seg["L"], seg["sel"]
         out["sel_gap"][r] = seg["sel_gap"]
         for name in ("o_far", "lse_far", "o_ret", "lse_ret", "o_loc", "lse_loc"):
             out[name][r] = seg[name]
     out["summ"] = summ
+    out["cbar"] = cbar
     return out
 
 
@@ -402,7 +462,7 @@ def _head_map(Hq, Hkv, head_map):
 
 
 def layer_forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, sel_mode=0,
-                  head_map=None):
+                  head_map=None, dipole=0):
     B, Hq, N, D = Q.shape
     Hkv = K.shape[1]
     hm = _head_map(Hq, Hkv, head_map)
@@ -413,7 +473,7 @@ def layer_forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=
             g = hm[h]
             f = forward(Q[b, h], K[b, g], V[b, g], a_q[b, h], a_k[b, g], qbar[b, h], sigma=sigma,
                         S=S, Ck=Ck, m=m, causal=causal, sel=None if sel is None else sel[b, h],
-                        sel_mode=sel_mode)
+                        sel_mode=sel_mode, dipole=dipole)
             O[b, h], LSE[b, h], SEL[b, h] = f["O"], f["LSE"], f["sel"]
     return O, LSE, SEL
 
