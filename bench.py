@@ -78,6 +78,12 @@ def work_model(w: wl.Workload):
         "k_merge": ("hbm", heads * nd * (8 + e) + part + heads * N * m * 4),
         "k_final_dq": ("hbm", heads * nd * (4 + e) + part),
         "k_final_dkv": ("hbm", heads * 4 * nd * 4 + kvh * 2 * nd * e),
+        # dipole correction (only with --dipole): covariances written once, merged by one GEMM per
+        # (head, plane), consumed once per query
+        "k_dipole_cov": ("hbm", kvh * SB * Ck * D * D * e + 2 * kvh * nd * e),
+        "k_dipole_merge_tc": ("tensor", 2.0 * heads * SB * Cq * Ck * D * D),
+        "k_dipole_merge": ("tensor", 2.0 * heads * SB * Cq * Ck * D * D),
+        "k_dipole_apply": ("hbm", heads * SB * Cq * D * D * e + heads * nd * (e + 8)),
     }
     return M
 
@@ -231,6 +237,8 @@ def main():
                     help="run the KV-head groups in this many sequential stages over one set of buffers "
                          "(0 = as few as keep the summaries under 64 GB)")
     ap.add_argument("--forward-only", action="store_true", help="time cluster + summarize + forward only")
+    ap.add_argument("--dipole", action="store_true",
+                    help="far field with the dipole correction instead of retrieval (sets m = 0, forward only)")
     ap.add_argument("--ref-rows", type=int, default=128, help="sampled queries for the oracle timing")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
@@ -241,6 +249,9 @@ def main():
     w = wl.WORKLOADS[args.workload]
     if args.m is not None:
         w = w.with_(m=args.m)
+    if args.dipole:
+        w = w.with_(m=0)
+        args.forward_only = True
     if args.heads is not None:
         w = w.with_(Hq=args.heads, Hkv=max(1, args.heads * w.Hkv // w.Hq))
     if args.impl == "reference":
@@ -280,7 +291,7 @@ def main():
         raise SystemExit("head staging needs B == 1 and a group count that divides the KV heads")
     hq, hkv = w.Hq // groups, w.Hkv // groups
     p = mb.make_params(B=w.B, Hq=hq, Hkv=hkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=w.m, n_blocks=w.S,
-                       dtype=w.dtype, kmeans_iters=w.T)
+                       dtype=w.dtype, kmeans_iters=w.T, dipole=int(args.dipole))
     buf = mb.MuseBuffers(p, backward=not args.forward_only)
     O_all = torch.empty_like(Q)
     dQ_all, dK_all, dV_all = (None, None, None) if args.forward_only else (torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V))
@@ -381,7 +392,7 @@ def main():
         else:
             ach, peak, unit = work / sec / 1e9, pk["hbm"], "GB/s"
         traffic = None
-        if w.name == "headline" and args.m is None and top in NCU_TRAFFIC_PER_HEAD:
+        if w.name == "headline" and w.m == 32 and top in NCU_TRAFFIC_PER_HEAD:
             traffic = NCU_TRAFFIC_PER_HEAD[top] * w.B * w.Hq    # one launch per step covers all heads
         roof.update(bound=bound, achieved=ach, peak=peak, unit=unit, frac=ach / peak, traffic=traffic,
                     peak_source=pk["source"] + (" (sustained bf16)" if bound == "tensor" else " (copy)"),
@@ -430,7 +441,7 @@ def main():
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype,
             "data": "synthetic",
             "config": dict(workload_config(w, args.gain), head_stages=groups,
-                           passes="cluster+summarize+forward" if args.forward_only else "cluster+summarize+forward+backward"),
+                           dipole=int(args.dipole), passes="cluster+summarize+forward" if args.forward_only else "cluster+summarize+forward+backward"),
             "clocks": clocks, "e2e": e2e,
             "gpu_launches": launches, "roofline": roof, "cpu_baseline": cpu, "kernels": kernels, "context": context}
     print(json.dumps(line))

@@ -73,7 +73,9 @@ typedef struct muse_params {
   uint64_t seed;                /* used by MUSE_INIT_STRIDED                                       */
   int32_t sel_mode;             /* MUSE_SEL_*: rank clusters by the Eq. 6 score per query, or by
                                    the accumulated log-mass per (query cluster, block)            */
-  int32_t dipole;               /* must be 0 (the dipole correction of Appendix B is not built)    */
+  int32_t dipole;               /* 0 off; 1: untilted, pre-merged dipole correction of the far field
+                                   (Appendix "Error Analysis", "Dipole Correction"); forward only,
+                                   requires m == 0 as in the paper                                   */
   int32_t agg_grad;             /* 1: differentiate the tilted aggregation weights; 0: constants   */
   const int32_t* head_map;      /* HOST [Hq] -> kv head, or NULL for h * Hkv / Hq                  */
 } muse_params_t;
@@ -95,8 +97,11 @@ MUSE_API int muse_workspace_bytes(const muse_params_t* p, size_t out[5]);
  *   off[3] kappa_lo  [e][D] ... and the bf16 rounding of the remainder (kappa = hi + lo);
  *                           fp32 mode: unused (same offset as off[4])
  *   off[4] nu        [e][D] fp32 (fp32 mode) or bf16 (bf16 mode)
- *   off[5], off[6]          K and V bucketed by (cluster, block), [B,Hkv,N,D] dtype */
-MUSE_API int muse_summaries_layout(const muse_params_t* p, size_t off[7]);
+ *   off[5], off[6]          K and V bucketed by (cluster, block), [B,Hkv,N,D] dtype
+ *   off[7] cbar             dipole == 1 only: merged dipole matrices Cbar = sum_j p(j) Cov_0j(v,k),
+ *                           [B,Hq,SB,Cq][D value dims][D key dims], fp32 (fp32 mode) or bf16; with
+ *                           dipole == 0 nothing is stored there (off[7] = end of the buffer) */
+MUSE_API int muse_summaries_layout(const muse_params_t* p, size_t off[8]);
 
 /* Lloyd k-means of the queries (per query head, Cq clusters) and keys (per kv head, Ck
  * clusters): T x (assign to argmin_c |c|^2 - 2 x.c, lowest index on ties; move each centre to

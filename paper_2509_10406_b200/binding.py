@@ -142,7 +142,7 @@ def muse_profile_report() -> dict:
 
 def muse_summaries_layout(p: MuseParams):
     """Byte offsets (mu, beta, kappa, kappa_lo, nu, K bucketed, V bucketed)."""
-    out = (ctypes.c_size_t * 7)()
+    out = (ctypes.c_size_t * 8)()
     _check(lib().muse_summaries_layout(ctypes.byref(p), out), "muse_summaries_layout")
     return tuple(int(x) for x in out)
 

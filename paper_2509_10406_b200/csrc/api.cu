@@ -19,7 +19,9 @@ int resolve(const muse_params_t* p, Dims* d) {
   if (p->n_blocks < 0 || p->k2 < 0) return MUSE_ERR_INVALID_ARG;
   if (p->D != 64 && p->D != 128) return MUSE_ERR_UNSUPPORTED;
   if (p->Hq > kMaxHeads || p->m > kMaxM || p->Cq > kMaxC || p->Ck > kMaxC) return MUSE_ERR_UNSUPPORTED;
-  if (p->k2 != 0 || p->dipole != 0) return MUSE_ERR_UNSUPPORTED;
+  if (p->dipole != 0 && p->dipole != 1) return MUSE_ERR_INVALID_ARG;
+  if (p->k2 != 0) return MUSE_ERR_UNSUPPORTED;
+  if (p->dipole != 0 && p->m != 0) return MUSE_ERR_UNSUPPORTED;      // the paper defines the dipole without retrieval
   int S = p->causal ? (p->n_blocks == 0 ? 8 : p->n_blocks) : 1;
   if (p->N % S != 0) return MUSE_ERR_INVALID_ARG;
   if ((long long)S * p->Cq > 32768 || (long long)S * p->Ck > 32768) return MUSE_ERR_UNSUPPORTED;
@@ -28,6 +30,7 @@ int resolve(const muse_params_t* p, Dims* d) {
   d->Cq = p->Cq; d->Ck = p->Ck; d->m = p->m;
   d->S = S; d->SB = p->causal ? S - 1 : 1; d->Bs = p->N / S;
   d->causal = p->causal ? 1 : 0; d->sel_mode = p->sel_mode; d->agg_grad = p->agg_grad ? 1 : 0;
+  d->dipole = p->dipole;
   d->sigma = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->D);
   for (int h = 0; h < kMaxHeads; ++h) d->hm.g[h] = 0;
   for (int h = 0; h < p->Hq; ++h) {
@@ -62,7 +65,7 @@ int muse_workspace_bytes(const muse_params_t* p, size_t out[5]) {
   if (out == nullptr) return MUSE_ERR_INVALID_ARG;
   size_t cq = lloyd_ws_bytes(d, d.B * d.Hq, d.Cq, 0), ck = lloyd_ws_bytes(d, d.B * d.Hkv, d.Ck, 1);
   out[0] = cq > ck ? cq : ck;
-  out[1] = summarize_ws_bytes(d);
+  out[1] = summarize_ws_bytes(d, p->dtype);
   out[2] = attn_fwd_ws_bytes(d, p->dtype);
   out[3] = attn_bwd_ws_bytes(d, p->dtype);
   out[4] = summ_layout(d, p->dtype).total;
@@ -70,13 +73,13 @@ int muse_workspace_bytes(const muse_params_t* p, size_t out[5]) {
   return MUSE_OK;
 }
 
-int muse_summaries_layout(const muse_params_t* p, size_t off[7]) {
+int muse_summaries_layout(const muse_params_t* p, size_t off[8]) {
   Dims d;
   int rc = resolve(p, &d);
   if (rc != MUSE_OK) return rc;
   if (off == nullptr) return MUSE_ERR_INVALID_ARG;
   SummLayout L = summ_layout(d, p->dtype);
-  off[0] = L.mu; off[1] = L.beta; off[2] = L.khi; off[3] = L.klo; off[4] = L.nu; off[5] = L.Kp; off[6] = L.Vp;
+  off[0] = L.mu; off[1] = L.beta; off[2] = L.khi; off[3] = L.klo; off[4] = L.nu; off[5] = L.Kp; off[6] = L.Vp; off[7] = L.cbar;
   return MUSE_OK;
 }
 
@@ -148,6 +151,7 @@ int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K, const vo
   int rc = resolve(p, &d);
   if (rc != MUSE_OK) return rc;
   if (!Q || !K || !V || !O || !LSE || !dO || !assign_q || !qbar || !off_k || !perm_k || !summaries || !dQ || !dK || !dV || !ws) return MUSE_ERR_INVALID_ARG;
+  if (d.dipole) return MUSE_ERR_UNSUPPORTED;       // no backward through the dipole correction
   if (d.m > 0 && d.SB > 0 && sel == nullptr) return MUSE_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(qbar) ||
       !aligned16(summaries) || !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;

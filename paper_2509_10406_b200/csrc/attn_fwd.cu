@@ -556,6 +556,10 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
           d, Q, qbar, w.off_q, w.perm_q, summ_ptrs(L, base), sel_in, sel, w.o_far, w.lse_far);
       MUSE_LAUNCH_OK();
     }
+    if (d.dipole) {
+      rc = dipole_apply(d, dtype, Q, qbar, w.off_q, w.perm_q, base + L.cbar, w.lse_far, w.o_far, st);
+      if (rc != MUSE_OK) return rc;
+    }
     if (d.m > 0) {
       RetIndex ri;
       rc = build_ret_index(d, sel, w.ret_scratch, &ri, st);

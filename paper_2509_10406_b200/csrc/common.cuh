@@ -22,6 +22,7 @@ struct Dims {
   int SB;       // stored summary planes: S-1 (causal) or 1
   int Bs;       // block size N / S
   int causal, sel_mode, agg_grad;
+  int dipole;   // 1: untilted pre-merged dipole correction of the far field (needs m == 0)
   float sigma;
   HeadMap hm;
 };
@@ -95,7 +96,14 @@ size_t lloyd_ws_bytes(const Dims& d, int problems, int C, int kind);
 int summarize(const Dims& d, int dtype, const void* K, const void* V, const int32_t* assign_k,
               const float* qbar, int32_t* off_k, int32_t* perm_k, void* summaries, void* ws,
               cudaStream_t st);
-size_t summarize_ws_bytes(const Dims& d);
+size_t summarize_ws_bytes(const Dims& d, int dtype);
+
+// dipole correction (dipole.cu): construction at summary time, consumption after the far field
+size_t dipole_ws_bytes(const Dims& d, int dtype);
+int dipole_build(const Dims& d, int dtype, const void* Kp, const void* Vp, const int32_t* off_k, const float* mu,
+                 void* cbar, void* ws, int* status, cudaStream_t st);
+int dipole_apply(const Dims& d, int dtype, const void* Q, const float* qbar, const int32_t* off_q, const int32_t* perm_q,
+                 const void* cbar, const float* lse_far, float* o_far, cudaStream_t st);
 
 // Byte offsets inside the caller's summaries buffer.  Per entry (b, h, plane, i, j):
 //   mu   fp32  accumulated log-mass            beta fp32  mu - sigma qbar_i . kappa  (so that the
@@ -103,7 +111,8 @@ size_t summarize_ws_bytes(const Dims& d);
 //   fp32 mode: kappa, nu fp32 [D]   (klo unused)
 //   bf16 mode: kappa = khi + klo, two bf16 planes [D] (tensor-core operands that keep ~16 bits
 //              of mantissa, so discrete top-m decisions match fp64); nu one bf16 plane [D]
-struct SummLayout { size_t mu, beta, khi, klo, nu, Kp, Vp, total; };
+//   cbar (dipole only): merged dipole matrices [B,Hq,SB,Cq][D value dims][D key dims], fp32 or bf16
+struct SummLayout { size_t mu, beta, khi, klo, nu, Kp, Vp, cbar, total; };
 SummLayout summ_layout(const Dims& d, int dtype);
 
 struct SummPtrs { float* mu; float* beta; void* khi; void* klo; void* nu; };

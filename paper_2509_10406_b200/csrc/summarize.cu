@@ -23,7 +23,8 @@ SummLayout summ_layout(const Dims& d, int dtype) {
   L.nu = dtype == MUSE_F32 ? L.klo : up(L.klo + ent * d.D * es);
   L.Kp = up(L.nu + ent * d.D * es);
   L.Vp = up(L.Kp + (size_t)d.B * d.Hkv * d.N * d.D * es);
-  L.total = up(L.Vp + (size_t)d.B * d.Hkv * d.N * d.D * es);
+  L.cbar = up(L.Vp + (size_t)d.B * d.Hkv * d.N * d.D * es);
+  L.total = up(L.cbar + (d.dipole ? (size_t)d.B * d.Hq * d.SB * d.Cq * d.D * d.D * es : 0));
   return L;
 }
 
@@ -168,6 +169,10 @@ k_summarize(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const i
 }
 
 template <class T, int D>
+static int summarize_planes(const Dims& d, int dtype, const T* Kp, const T* Vp, const int32_t* off_k, const float* qbar,
+                            const SummLayout& L, char* base, int32_t* status, cudaStream_t st);
+
+template <class T, int D>
 static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const int32_t* assign_k,
                        const float* qbar, int32_t* off_k, int32_t* perm_k, void* summaries, void* ws,
                        cudaStream_t st) {
@@ -186,11 +191,19 @@ static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const i
   k_gather_rows<T><<<gg, 256, 0, st>>>(V, perm_k, d.N, D, Vp);
   MUSE_LAUNCH_OK();
   if (d.SB == 0) return MUSE_OK;
-  if (summarize_tc_supported(d, dtype) && getenv("MUSE_SUMM_FWD_SIMT") == nullptr) {
-    int32_t* status = (int32_t*)ws + sort_ws_elems(d.N, d.Ck * d.S) * (size_t)pk;      // 64 words after the sort scratch
-    MUSE_CUDA_OK(cudaMemsetAsync(status, 0, 64 * sizeof(int32_t), st));
+  Arena ar(ws);
+  int32_t* status = ar.take<int32_t>(sort_ws_elems(d.N, d.Ck * d.S) * (size_t)pk + 64) + sort_ws_elems(d.N, d.Ck * d.S) * (size_t)pk;
+  MUSE_CUDA_OK(cudaMemsetAsync(status, 0, 64 * sizeof(int32_t), st));     // 64 words after the sort scratch
+  rc = summarize_planes<T, D>(d, dtype, Kp, Vp, off_k, qbar, L, base, status, st);
+  if (rc != MUSE_OK || !d.dipole) return rc;
+  return dipole_build(d, dtype, Kp, Vp, off_k, summ_ptrs(L, base).mu, base + L.cbar, (char*)ws + ar.used, status, st);
+}
+
+template <class T, int D>
+static int summarize_planes(const Dims& d, int dtype, const T* Kp, const T* Vp, const int32_t* off_k, const float* qbar,
+                            const SummLayout& L, char* base, int32_t* status, cudaStream_t st) {
+  if (summarize_tc_supported(d, dtype) && getenv("MUSE_SUMM_FWD_SIMT") == nullptr)
     return summarize_tc(d, Kp, Vp, off_k, qbar, summ_ptrs(L, base), status, st);
-  }
   const size_t smem = (size_t)(kSumI * (D + 4) + kSumKC * (2 * D + 4) + kSumI * (kSumKC + 1)) * sizeof(float);
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid(d.Ck, cdiv(d.Cq, kSumI), d.B * d.Hq);
@@ -200,10 +213,10 @@ static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const i
   return MUSE_OK;
 }
 
-size_t summarize_ws_bytes(const Dims& d) {
+size_t summarize_ws_bytes(const Dims& d, int dtype) {
   Arena ar(nullptr);
   ar.take<int32_t>((size_t)d.B * d.Hkv * sort_ws_elems(d.N, d.Ck * d.S) + 64);
-  return ar.used;
+  return ar.used + dipole_ws_bytes(d, dtype);
 }
 
 int summarize(const Dims& d, int dtype, const void* K, const void* V, const int32_t* assign_k,

@@ -38,13 +38,13 @@ def test_workspace_sizes_and_layout(mb):
     assert sizes[4] >= ent * (3 * 128 * 2 + 8) + 2 * 16 * 65536 * 128 * 2
     off = mb.muse_summaries_layout(p)
     assert off[0] == 0 and off[1] >= ent * 4 and off[3] - off[2] >= ent * 128 * 2 and all(o % 256 == 0 for o in off)
-    assert len(off) == 7 and list(off) == sorted(off)
+    assert len(off) == 8 and list(off) == sorted(off)
     assert all(s % 256 == 0 for s in sizes)
 
 
 @pytest.mark.parametrize("kw,code", [
     (dict(D=96), -2), (dict(m=2000), -1), (dict(N=1001), -1), (dict(Cq=0), -1), (dict(k2=1), -2),
-    (dict(dipole=1), -2), (dict(Hq=3, Hkv=2), -1), (dict(m=65, Ck=128), -2), (dict(Ck=8192, N=16384), -2),
+    (dict(dipole=1), -2), (dict(dipole=2), -1), (dict(Hq=3, Hkv=2), -1), (dict(m=65, Ck=128), -2), (dict(Ck=8192, N=16384), -2),
 ])
 def test_invalid_parameters_are_rejected_on_the_host(mb, kw, code):
     args = dict(B=1, Hq=2, Hkv=2, N=1024, D=64, Cq=8, Ck=16, m=4)

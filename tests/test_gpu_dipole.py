@@ -1,0 +1,83 @@
+"""GPU parity for the dipole correction of the far field (untilted, pre-merged, m = 0): merged
+matrices and forward outputs against the fp64 oracle, teacher-forced clustering.  Tolerance:
+max-abs error relative to the oracle tensor's max-abs <= 1e-4 (fp32 mode), 2e-2 (bf16 mode)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import muse_oracle as orc
+from tests.gpu_util import Case, to_dev, to_np, tol, rel_err
+from tests.test_gpu_cluster import CASES
+
+pytestmark = pytest.mark.gpu
+
+DIPOLE_CASES = {
+    "tiny_f32": (CASES["tiny"].with_(m=0), True),
+    "tiny_f32_noncausal": (CASES["tiny"].with_(m=0), False),
+    "gqa_bf16_d64": (CASES["gqa_bf16"].with_(B=1, Hq=2, Hkv=1, m=0), True),            # tensor merge, D = 64, Cq < 128
+    "d128_bf16": (CASES["d128"].with_(m=0), True),                                      # tensor merge, ragged Cq = 24
+    "d128_bf16_two_halves": (CASES["d128"].with_(m=0, Hq=1, Hkv=1, N=2048, Cq=160, Ck=64), True),
+    "d128_f32_odd_ck": (CASES["d128"].with_(dtype="f32", m=0, Hq=1, Hkv=1, N=1000, Cq=8, Ck=24, S=4), True),
+}
+
+
+def _cbar(mb, p, buf):
+    off = mb.muse_summaries_layout(p)
+    n = p.B * p.Hq * p.SB * p.Cq * p.D * p.D
+    if p.dtype == mb.MUSE_F32:
+        t = buf.summaries[off[7]:off[7] + 4 * n].view(torch.float32)
+    else:
+        t = buf.summaries[off[7]:off[7] + 2 * n].view(torch.bfloat16).float()
+    return to_np(t).reshape(p.B, p.Hq, p.SB, p.Cq, p.D, p.D)
+
+
+@pytest.mark.parametrize("name", list(DIPOLE_CASES))
+@pytest.mark.parametrize("gain", [1.0, 128.0])
+def test_dipole_forward_matches_oracle(name, gain):
+    from paper_2509_10406_b200 import binding as mb
+    w, causal = DIPOLE_CASES[name]
+    c = Case(w, gain=gain)
+    qbar32 = c.qbar.astype(np.float32)
+    p = c.params(dipole=1, causal=causal)
+    buf = mb.MuseBuffers(p, backward=False)
+    Q, K, V, _ = c.dev()
+    a_q, a_k, qb = to_dev(c.a_q, "i"), to_dev(c.a_k, "i"), to_dev(qbar32, "f32")
+    mb.muse_summarize(p, K, V, a_k, qb, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
+    mb.muse_attn_fwd(p, Q, K, V, a_q, qb, buf.off_k, buf.perm_k, buf.summaries, None, buf.O, buf.LSE, buf.sel, buf.ws)
+    torch.cuda.synchronize()
+    assert int(buf.ws[:4].view(torch.int32)[0]) == 0
+    O, L, cb = to_np(buf.O), to_np(buf.LSE), _cbar(mb, p, buf)
+    t = tol(w.dtype)
+    S = w.S if causal else 1
+    moved = 0.0
+    for b in range(w.B):
+        for h in range(w.Hq):
+            g = c.hm[h]
+            kw = dict(sigma=c.sigma, S=w.S, Ck=w.Ck, m=0, causal=causal)
+            f1 = orc.forward(c.Q[b, h], c.K[b, g], c.V[b, g], c.a_q[b, h], c.a_k[b, g], qbar32[b, h].astype(np.float64), dipole=1, **kw)
+            f0 = orc.forward(c.Q[b, h], c.K[b, g], c.V[b, g], c.a_q[b, h], c.a_k[b, g], qbar32[b, h].astype(np.float64),
+                             summ=f1["summ"], **kw)
+            ref = f1["cbar"][1:] if causal else f1["cbar"]
+            assert ref.shape == cb[b, h].shape and len(ref) == (S - 1 if causal else 1)
+            # the matrices only matter for query clusters that own queries in the plane's block
+            assert rel_err(cb[b, h], ref) <= t
+            assert rel_err(O[b, h], f1["O"]) <= t
+            assert np.abs(L[b, h] - f1["LSE"]).max() <= 1e-3 * max(1.0, np.abs(f1["LSE"]).max())
+            moved = max(moved, rel_err(f0["O"], f1["O"]))
+            # the GPU result must be closer to the oracle with the correction than to the one without,
+            # wherever the correction is larger than the tolerance
+            if rel_err(f0["O"], f1["O"]) > 4 * t:
+                assert rel_err(O[b, h], f1["O"]) < rel_err(O[b, h], f0["O"])
+    assert moved > 0.0
+
+
+def test_dipole_argument_rules():
+    from paper_2509_10406_b200 import binding as mb
+    w = CASES["tiny"]
+    with pytest.raises(mb.MuseError):
+        mb.muse_workspace_bytes(mb.make_params(B=1, Hq=1, Hkv=1, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=2, dipole=1))
+    p0 = mb.make_params(B=1, Hq=1, Hkv=1, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=0, dtype="f32")
+    p1 = mb.make_params(B=1, Hq=1, Hkv=1, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=0, dtype="f32", dipole=1)
+    s0, s1 = mb.muse_workspace_bytes(p0), mb.muse_workspace_bytes(p1)
+    assert s1[4] >= s0[4] + 7 * w.Cq * w.D * w.D * 4 and s1[1] > s0[1]
+    assert mb.muse_summaries_layout(p0)[7] == s0[4]
