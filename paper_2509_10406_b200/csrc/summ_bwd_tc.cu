@@ -20,11 +20,13 @@ namespace muse {
 typedef __nv_bfloat16 bf16;
 
 namespace sb {
-constexpr int D = 128, TI = 128, NU = 64;
+constexpr int D = 128, TI = 128, NU = 64, THREADS = 256;
 constexpr int kTile = TI * D * 2;              // 32 KB
 constexpr int kKeys = NU * D * 2;              // 16 KB
-constexpr int oQhi = 0, oQlo = oQhi + kTile, oDka = oQlo + kTile, oDnu = oDka + kTile;
-constexpr int oK = oDnu + kTile, oV = oK + kKeys, oW = oV + kKeys, oWc = oW + TI * NU * 2;
+// The low half of the centroid tile is only needed for the tilt logits, which do not depend on
+// the plane: once they are in TMEM its space serves as the second dkappa buffer.
+constexpr int oQhi = 0, oQlo = oQhi + kTile, oDka0 = oQlo + kTile, oDnu0 = oDka0 + kTile, oDnu1 = oDnu0 + kTile;
+constexpr int oK = oDnu1 + kTile, oV = oK + kKeys, oW = oV + kKeys, oWc = oW + TI * NU * 2;
 constexpr int total = oWc + TI * NU * 2 + 1024;
 constexpr uint32_t cL = 0, cX1 = 64, cX2 = 128, cDK = 192, cDV = 256;
 }  // namespace sb
@@ -32,7 +34,7 @@ constexpr uint32_t cL = 0, cX1 = 64, cX2 = 128, cDK = 192, cDV = 256;
 // 2-D tensor map over a bf16 matrix with an arbitrary row pitch (bytes), 128B swizzle, box [box_rows][64]
 int make_tmap_bf16_pitched(void* out_map, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows);
 
-__global__ void __launch_bounds__(128, 1)
+__global__ void __launch_bounds__(sb::THREADS, 1)
 k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_constant__ CUtensorMap tm_dnu,
               const __grid_constant__ CUtensorMap tm_K, const __grid_constant__ CUtensorMap tm_V,
               const int32_t* __restrict__ off_k, const int32_t* __restrict__ off_q, const float* __restrict__ qbar,
@@ -40,27 +42,29 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
               float* __restrict__ dV_perm, int* __restrict__ status) {
   using namespace sb;
   extern __shared__ __align__(1024) unsigned char sm_raw[];
-  __shared__ uint64_t bar_g, bar_kv, bar1, bar2;
+  __shared__ uint64_t bar_g[2], bar_kv, bar_l, bar1, bar2;
   __shared__ uint32_t tbase_s;
   const int j = blockIdx.x, pq = blockIdx.y;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, wg = tid >> 7, L = tid & 127;
   const int32_t* ok_ = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const int32_t* oq = off_q + (size_t)pq * (dm.S * dm.Cq + 1);
   const int kbeg = ok_[0];
   if (kbeg >= ok_[dm.SB]) return;                       // no key of this cluster is ever summarised
   unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
   if (warp == 0) tc::tmem_alloc(&tbase_s, 512);
-  if (tid == 0) { tc::mbar_init(&bar_g, 1); tc::mbar_init(&bar_kv, 1); tc::mbar_init(&bar1, 1); tc::mbar_init(&bar2, 1); tc::mbar_init_fence(); }
+  if (tid == 0) {
+    tc::mbar_init(&bar_g[0], 1); tc::mbar_init(&bar_g[1], 1); tc::mbar_init(&bar_kv, 1); tc::mbar_init(&bar_l, 1);
+    tc::mbar_init(&bar1, 1); tc::mbar_init(&bar2, 1); tc::mbar_init_fence();
+  }
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
-  const uint32_t tbase = tbase_s, tlane = tbase + ((uint32_t)(warp * 32) << 16);
-  uint32_t ph_g = 0, ph_kv = 0, ph1 = 0, ph2 = 0;
+  const uint32_t tbase = tbase_s, tlane = tbase + ((uint32_t)((warp & 3) * 32) << 16);
+  uint32_t ph_g[2] = {0, 0}, ph_kv = 0, ph_l = 0, ph1 = 0, ph2 = 0;
   bool ok = true;
-  const uint32_t aQhi = tc::smem_u32(sm + oQhi), aQlo = tc::smem_u32(sm + oQlo), aDka = tc::smem_u32(sm + oDka),
-                 aDnu = tc::smem_u32(sm + oDnu), aK = tc::smem_u32(sm + oK), aV = tc::smem_u32(sm + oV),
-                 aW = tc::smem_u32(sm + oW), aWc = tc::smem_u32(sm + oWc);
+  const uint32_t aQhi = tc::smem_u32(sm + oQhi), aQlo = tc::smem_u32(sm + oQlo), aK = tc::smem_u32(sm + oK),
+                 aV = tc::smem_u32(sm + oV), aW = tc::smem_u32(sm + oW), aWc = tc::smem_u32(sm + oWc);
 
   const int kvis = ok_[dm.SB];
   for (int c0 = kbeg; c0 < kvis && ok; c0 += NU) {        // 64 keys of the cluster at a time (usually one chunk)
@@ -71,20 +75,34 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
       tc::tma_load_2d(sm + oK, &tm_K, 0, row, &bar_kv); tc::tma_load_2d(sm + oK + NU * 128, &tm_K, 64, row, &bar_kv);
       tc::tma_load_2d(sm + oV, &tm_V, 0, row, &bar_kv); tc::tma_load_2d(sm + oV + NU * 128, &tm_V, 64, row, &bar_kv);
     }
+    int pl0 = 0;                                          // planes [pl0, SB) see this chunk (bucket ends grow with the plane)
+    while (pl0 < dm.SB && ok_[pl0 + 1] <= c0) ++pl0;
     if (!tc::mbar_wait(&bar_kv, ph_kv)) ok = false;
     ph_kv ^= 1;
     bool started = false;                                 // dK^T / dV^T accumulate in TMEM over all (i tile, plane)
     for (int i0 = 0; i0 < dm.Cq && ok; i0 += TI) {
-      // sigma * qbar tile as bf16 hi + lo (thread = row)
-      __syncthreads();
+      const int i = i0 + L;
+      const bool in_range = i < dm.Cq;
+      const int ic = in_range ? i : 0;
+      auto issue_grad = [&](int pl, int buf) {            // thread 0: both gradient tiles of (plane, j, i0..i0+127)
+        tc::mbar_expect_tx(&bar_g[buf], 2 * kTile);
+        const int row = (int)((((size_t)pq * dm.SB + pl) * dm.Ck + j) * dm.Cq + i0);
+        unsigned char* dka = sm + (buf ? oQlo : oDka0);
+        unsigned char* dnu = sm + (buf ? oDnu1 : oDnu0);
+        tc::tma_load_2d(dka, &tm_dka, 0, row, &bar_g[buf]); tc::tma_load_2d(dka + TI * 128, &tm_dka, 64, row, &bar_g[buf]);
+        tc::tma_load_2d(dnu, &tm_dnu, 0, row, &bar_g[buf]); tc::tma_load_2d(dnu + TI * 128, &tm_dnu, 64, row, &bar_g[buf]);
+      };
+      __syncthreads();                                    // every MMA that read the centroid tiles has completed (bar2 waited)
+      if (tid == 0 && pl0 < dm.SB) issue_grad(pl0, 0);
+      // sigma * qbar tile as bf16 hi + lo (thread = row, warpgroup = half of the 16-byte chunks)
       {
-        const int i = i0 + tid;
-        const float* src = qbar + ((size_t)pq * dm.Cq + (i < dm.Cq ? i : 0)) * D;
+        const float* src = qbar + ((size_t)pq * dm.Cq + ic) * D;
 #pragma unroll
-        for (int ck = 0; ck < D / 8; ++ck) {
+        for (int c8 = 0; c8 < D / 16; ++c8) {
+          const int ck = wg * (D / 16) + c8;
           uint32_t wh[4], wl[4];
-          const float4 f0 = i < dm.Cq ? ld4(src + ck * 8) : make_float4(0.f, 0.f, 0.f, 0.f);
-          const float4 f1 = i < dm.Cq ? ld4(src + ck * 8 + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+          const float4 f0 = in_range ? ld4(src + ck * 8) : make_float4(0.f, 0.f, 0.f, 0.f);
+          const float4 f1 = in_range ? ld4(src + ck * 8 + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
           const float x[8] = {f0.x * dm.sigma, f0.y * dm.sigma, f0.z * dm.sigma, f0.w * dm.sigma,
                               f1.x * dm.sigma, f1.y * dm.sigma, f1.z * dm.sigma, f1.w * dm.sigma};
 #pragma unroll
@@ -93,34 +111,66 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
             __nv_bfloat162 ll = __floats2bfloat162_rn(x[2 * e] - __low2float(hh), x[2 * e + 1] - __high2float(hh));
             wh[e] = *reinterpret_cast<uint32_t*>(&hh); wl[e] = *reinterpret_cast<uint32_t*>(&ll);
           }
-          const uint32_t off = (ck >> 3) * TI * 128 + tc::sw128_off(tid, ck & 7);
+          const uint32_t off = (ck >> 3) * TI * 128 + tc::sw128_off(L, ck & 7);
           *reinterpret_cast<uint4*>(sm + oQhi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
           *reinterpret_cast<uint4*>(sm + oQlo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
         }
       }
-      for (int pl = 0; pl < dm.SB && ok; ++pl) {
-        const int kend = ok_[pl + 1];
-        if (kend <= c0) continue;                         // this plane does not see the chunk
-        const int nk = min(NU, kend - c0);
-        const int i = i0 + tid, blk = dm.causal ? pl + 1 : 0;
-        const size_t gent = (((size_t)pq * dm.SB + pl) * dm.Ck + j) * dm.Cq + (i < dm.Cq ? i : 0);     // gradients: [plane][j][i]
-        const size_t ent = (((size_t)pq * dm.SB + pl) * dm.Cq + (i < dm.Cq ? i : 0)) * dm.Ck + j;      // summaries: [plane][i][j]
-        const bool live = i < dm.Cq && oq[(size_t)blk * dm.Cq + i + 1] > oq[(size_t)blk * dm.Cq + i];
-        const float mu_i = live ? mu[ent] : 0.f, dS_i = live ? dS[gent] : 0.f;
-        __syncthreads();                                  // previous users of the gradient and w tiles are done
-        if (tid == 0) {
-          tc::mbar_expect_tx(&bar_g, 2 * kTile);
-          const int row = (int)((((size_t)pq * dm.SB + pl) * dm.Ck + j) * dm.Cq + i0);
-          tc::tma_load_2d(sm + oDka, &tm_dka, 0, row, &bar_g); tc::tma_load_2d(sm + oDka + TI * 128, &tm_dka, 64, row, &bar_g);
-          tc::tma_load_2d(sm + oDnu, &tm_dnu, 0, row, &bar_g); tc::tma_load_2d(sm + oDnu + TI * 128, &tm_dnu, 64, row, &bar_g);
+      // which planes hold a non-empty segment of query cluster i (others were never written by the far-field pass)
+      uint32_t livemask = 0u;
+      for (int pl = pl0; pl < dm.SB; ++pl) {
+        const int blk = dm.causal ? pl + 1 : 0;
+        if (in_range && oq[(size_t)blk * dm.Cq + i + 1] > oq[(size_t)blk * dm.Cq + i]) livemask |= 1u << pl;
+      }
+      tc::fence_async_smem();
+      tc::fence_before_sync();
+      __syncthreads();
+      // tilt logits l_iu = sigma qbar_i . k_u, the same for every plane: once per centroid tile
+      if (tid == 0) {
+        tc::fence_after_sync();
+        const uint32_t idesc = tc::idesc_bf16(TI, NU, 0, 0);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks)
+          tc::mma_bf16_ss(tbase + cL, tc::smem_desc_sw128(aQhi + (ks / 4) * TI * 128 + (ks % 4) * 32, 16, 1024),
+                          tc::smem_desc_sw128(aK + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks)
+          tc::mma_bf16_ss(tbase + cL, tc::smem_desc_sw128(aQlo + (ks / 4) * TI * 128 + (ks % 4) * 32, 16, 1024),
+                          tc::smem_desc_sw128(aK + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, 1);
+        tc::mma_commit(&bar_l);
+      }
+      __syncwarp();
+      if (!tc::mbar_wait(&bar_l, ph_l)) ok = false;       // from here on the low tile's space is free
+      ph_l ^= 1;
+      tc::fence_after_sync();
+      float lg[32];
+      tc::tmem_ld32(tlane + cL + 32 * wg, lg);            // this thread's logits: row i, keys 32 wg .. 32 wg + 31
+      // per-plane scalars, loaded one plane ahead
+      auto ent_of = [&](int pl) { return (((size_t)pq * dm.SB + pl) * dm.Cq + ic) * dm.Ck + j; };        // summaries: [plane][i][j]
+      auto gent_of = [&](int pl) { return (((size_t)pq * dm.SB + pl) * dm.Ck + j) * dm.Cq + ic; };      // gradients: [plane][j][i]
+      float mu_n = 0.f, dS_n = 0.f;
+      if (pl0 < dm.SB && ((livemask >> pl0) & 1u)) { mu_n = mu[ent_of(pl0)]; dS_n = dS[gent_of(pl0)]; }
+      for (int pl = pl0, k = 0; pl < dm.SB && ok; ++pl, ++k) {
+        const int buf = k & 1;
+        const int nk = min(NU, ok_[pl + 1] - c0);
+        const bool live = (livemask >> pl) & 1u;
+        const float mu_i = mu_n, dS_i = dS_n;
+        if (k > 0) {                                      // the MMAs of the previous plane are done with the other buffer and with W / Wc
+          if (!tc::mbar_wait(&bar2, ph2)) ok = false;
+          ph2 ^= 1;
+          tc::fence_after_sync();
         }
-        if (!tc::mbar_wait(&bar_g, ph_g)) ok = false;
-        ph_g ^= 1;
+        if (tid == 0 && pl + 1 < dm.SB && ok) issue_grad(pl + 1, buf ^ 1);
+        if (pl + 1 < dm.SB && ((livemask >> (pl + 1)) & 1u)) { mu_n = mu[ent_of(pl + 1)]; dS_n = dS[gent_of(pl + 1)]; }
+        if (!tc::mbar_wait(&bar_g[buf], ph_g[buf])) ok = false;
+        ph_g[buf] ^= 1;
+        const int oDka = buf ? oQlo : oDka0, oDnu = buf ? oDnu1 : oDnu0;
         // rows of query clusters whose segment is empty (or beyond Cq) were never written: clear them
         if (!live) {
 #pragma unroll
-          for (int ck = 0; ck < D / 8; ++ck) {
-            const uint32_t off = (ck >> 3) * TI * 128 + tc::sw128_off(tid, ck & 7);
+          for (int c8 = 0; c8 < D / 16; ++c8) {
+            const int ck = wg * (D / 16) + c8;
+            const uint32_t off = (ck >> 3) * TI * 128 + tc::sw128_off(L, ck & 7);
             *reinterpret_cast<uint4*>(sm + oDka + off) = make_uint4(0u, 0u, 0u, 0u);
             *reinterpret_cast<uint4*>(sm + oDnu + off) = make_uint4(0u, 0u, 0u, 0u);
           }
@@ -128,17 +178,10 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         tc::fence_async_smem();
         tc::fence_before_sync();
         __syncthreads();
+        const uint32_t aDka = tc::smem_u32(sm + oDka), aDnu = tc::smem_u32(sm + oDnu);
         if (tid == 0) {
           tc::fence_after_sync();
           const uint32_t idesc = tc::idesc_bf16(TI, NU, 0, 0);
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks)
-            tc::mma_bf16_ss(tbase + cL, tc::smem_desc_sw128(aQhi + (ks / 4) * TI * 128 + (ks % 4) * 32, 16, 1024),
-                            tc::smem_desc_sw128(aK + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks)
-            tc::mma_bf16_ss(tbase + cL, tc::smem_desc_sw128(aQlo + (ks / 4) * TI * 128 + (ks % 4) * 32, 16, 1024),
-                            tc::smem_desc_sw128(aK + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, 1);
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks)
             tc::mma_bf16_ss(tbase + cX1, tc::smem_desc_sw128(aDka + (ks / 4) * TI * 128 + (ks % 4) * 32, 16, 1024),
@@ -153,25 +196,23 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         if (!tc::mbar_wait(&bar1, ph1)) ok = false;
         ph1 ^= 1;
         tc::fence_after_sync();
-#pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-          float l[32], x1[32], x2[32];
-          tc::tmem_ld32(tlane + cL + 32 * hh, l);
-          tc::tmem_ld32(tlane + cX1 + 32 * hh, x1);
-          tc::tmem_ld32(tlane + cX2 + 32 * hh, x2);
+        {
+          float x1[32], x2[32];
+          tc::tmem_ld32(tlane + cX1 + 32 * wg, x1);
+          tc::tmem_ld32(tlane + cX2 + 32 * wg, x2);
           uint32_t ww[16], wc[16];
 #pragma unroll
           for (int c = 0; c < 32; c += 2) {
             float w0 = 0.f, w1 = 0.f, c0_ = 0.f, c1_ = 0.f;
-            if (live && 32 * hh + c < nk) { w0 = __expf(l[c] - mu_i); c0_ = w0 * (dS_i + x1[c] + x2[c]); }
-            if (live && 32 * hh + c + 1 < nk) { w1 = __expf(l[c + 1] - mu_i); c1_ = w1 * (dS_i + x1[c + 1] + x2[c + 1]); }
+            if (live && 32 * wg + c < nk) { w0 = __expf(lg[c] - mu_i); c0_ = w0 * (dS_i + x1[c] + x2[c]); }
+            if (live && 32 * wg + c + 1 < nk) { w1 = __expf(lg[c + 1] - mu_i); c1_ = w1 * (dS_i + x1[c + 1] + x2[c + 1]); }
             __nv_bfloat162 a = __floats2bfloat162_rn(w0, w1), b = __floats2bfloat162_rn(c0_, c1_);
             ww[c >> 1] = *reinterpret_cast<uint32_t*>(&a); wc[c >> 1] = *reinterpret_cast<uint32_t*>(&b);
           }
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
-            *reinterpret_cast<uint4*>(sm + oW + tc::sw128_off(tid, 4 * hh + ch)) = make_uint4(ww[4 * ch], ww[4 * ch + 1], ww[4 * ch + 2], ww[4 * ch + 3]);
-            *reinterpret_cast<uint4*>(sm + oWc + tc::sw128_off(tid, 4 * hh + ch)) = make_uint4(wc[4 * ch], wc[4 * ch + 1], wc[4 * ch + 2], wc[4 * ch + 3]);
+            *reinterpret_cast<uint4*>(sm + oW + tc::sw128_off(L, 4 * wg + ch)) = make_uint4(ww[4 * ch], ww[4 * ch + 1], ww[4 * ch + 2], ww[4 * ch + 3]);
+            *reinterpret_cast<uint4*>(sm + oWc + tc::sw128_off(L, 4 * wg + ch)) = make_uint4(wc[4 * ch], wc[4 * ch + 1], wc[4 * ch + 2], wc[4 * ch + 3]);
           }
         }
         tc::fence_async_smem();
@@ -198,23 +239,24 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         }
         started = true;
         __syncwarp();
+      }
+      if (pl0 < dm.SB) {                                  // last plane's MMAs
         if (!tc::mbar_wait(&bar2, ph2)) ok = false;
         ph2 ^= 1;
         tc::fence_after_sync();
       }
     }
-    // read-out once per key chunk: thread = d, columns = keys; add into the fp32 accumulators
+    // read-out once per key chunk: thread = d, warpgroup = half of the keys; add into the fp32 accumulators
     const int nkc = min(NU, kvis - c0);
-#pragma unroll
-    for (int hh = 0; hh < 2; ++hh) {
+    {
       float a[32], b[32];
-      tc::tmem_ld32(tlane + cDK + 32 * hh, a);
-      tc::tmem_ld32(tlane + cDV + 32 * hh, b);
+      tc::tmem_ld32(tlane + cDK + 32 * wg, a);
+      tc::tmem_ld32(tlane + cDV + 32 * wg, b);
       if (ok && started) {
 #pragma unroll
         for (int u = 0; u < 32; ++u) {
-          if (32 * hh + u < nkc) {
-            const size_t at = ((size_t)pq * dm.N + c0 + 32 * hh + u) * D + tid;
+          if (32 * wg + u < nkc) {
+            const size_t at = ((size_t)pq * dm.N + c0 + 32 * wg + u) * D + L;
             dK_perm[at] += a[u];
             dV_perm[at] += b[u];
           }
@@ -247,7 +289,7 @@ int summ_bwd_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* of
   if (rc != MUSE_OK) return rc;
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, sb::total));
   prof_mark("k_summ_bwd_tc", st);
-  k_summ_bwd_tc<<<dim3(d.Ck, d.B * d.Hq), 128, sb::total, st>>>(d, tdka, tdnu, tK, tV, off_k, off_q, qbar, mu, dS, dK_perm,
+  k_summ_bwd_tc<<<dim3(d.Ck, d.B * d.Hq), sb::THREADS, sb::total, st>>>(d, tdka, tdnu, tK, tV, off_k, off_q, qbar, mu, dS, dK_perm,
                                                                 dV_perm, status);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
