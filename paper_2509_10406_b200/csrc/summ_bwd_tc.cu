@@ -67,6 +67,13 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
                  aV = tc::smem_u32(sm + oV), aW = tc::smem_u32(sm + oW), aWc = tc::smem_u32(sm + oWc);
 
   const int kvis = ok_[dm.SB];
+#ifdef MUSE_PHASE_CLOCKS
+  long long pc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  long long t_ = clock64();
+#define PCLK(k) { long long n_ = clock64(); pc[k] += n_ - t_; t_ = n_; }
+#else
+#define PCLK(k)
+#endif
   for (int c0 = kbeg; c0 < kvis && ok; c0 += NU) {        // 64 keys of the cluster at a time (usually one chunk)
     __syncthreads();
     if (tid == 0) {
@@ -92,6 +99,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         tc::tma_load_2d(dka, &tm_dka, 0, row, &bar_g[buf]); tc::tma_load_2d(dka + TI * 128, &tm_dka, 64, row, &bar_g[buf]);
         tc::tma_load_2d(dnu, &tm_dnu, 0, row, &bar_g[buf]); tc::tma_load_2d(dnu + TI * 128, &tm_dnu, 64, row, &bar_g[buf]);
       };
+      PCLK(7)
       __syncthreads();                                    // every MMA that read the centroid tiles has completed (bar2 waited)
       if (tid == 0 && pl0 < dm.SB) issue_grad(pl0, 0);
       // sigma * qbar tile as bf16 hi + lo (thread = row, warpgroup = half of the 16-byte chunks)
@@ -143,6 +151,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
       if (!tc::mbar_wait(&bar_l, ph_l)) ok = false;       // from here on the low tile's space is free
       ph_l ^= 1;
       tc::fence_after_sync();
+      PCLK(0)
       float lg[32];
       tc::tmem_ld32(tlane + cL + 32 * wg, lg);            // this thread's logits: row i, keys 32 wg .. 32 wg + 31
       // per-plane scalars, loaded one plane ahead
@@ -160,10 +169,12 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
           ph2 ^= 1;
           tc::fence_after_sync();
         }
+        PCLK(1)
         if (tid == 0 && pl + 1 < dm.SB && ok) issue_grad(pl + 1, buf ^ 1);
         if (pl + 1 < dm.SB && ((livemask >> (pl + 1)) & 1u)) { mu_n = mu[ent_of(pl + 1)]; dS_n = dS[gent_of(pl + 1)]; }
         if (!tc::mbar_wait(&bar_g[buf], ph_g[buf])) ok = false;
         ph_g[buf] ^= 1;
+        PCLK(2)
         const int oDka = buf ? oQlo : oDka0, oDnu = buf ? oDnu1 : oDnu0;
         // rows of query clusters whose segment is empty (or beyond Cq) were never written: clear them
         if (!live) {
@@ -196,6 +207,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         if (!tc::mbar_wait(&bar1, ph1)) ok = false;
         ph1 ^= 1;
         tc::fence_after_sync();
+        PCLK(3)
         {
           float x1[32], x2[32];
           tc::tmem_ld32(tlane + cX1 + 32 * wg, x1);
@@ -239,6 +251,10 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         }
         started = true;
         __syncwarp();
+        PCLK(4)
+#ifdef MUSE_PHASE_CLOCKS
+        pc[6] += 1;
+#endif
       }
       if (pl0 < dm.SB) {                                  // last plane's MMAs
         if (!tc::mbar_wait(&bar2, ph2)) ok = false;
@@ -246,6 +262,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         tc::fence_after_sync();
       }
     }
+    PCLK(5)
     // read-out once per key chunk: thread = d, warpgroup = half of the keys; add into the fp32 accumulators
     const int nkc = min(NU, kvis - c0);
     {
@@ -268,6 +285,9 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tbase, 512);
+#ifdef MUSE_PHASE_CLOCKS
+  if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 0) for (int k = 0; k < 8; ++k) status[48 + k] = (int)pc[k];
+#endif
   if (!ok && tid == 0) atomicExch(status, 5);
 }
 

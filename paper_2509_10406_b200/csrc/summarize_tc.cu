@@ -8,7 +8,8 @@
 //   U   = W [K | V]             tcgen05 (keys contracted), folded into the accumulators with the
 //                               online-softmax rescale
 // After each bucket the normalised snapshot (mu, beta, kappa hi/lo, nu) of plane = bucket index
-// is staged in shared memory and leaves in coalesced 256-byte rows.
+// is staged in shared memory as three swizzled tiles that leave by TMA stores while the next
+// plane is being computed.
 #include <cuda.h>
 #include "common.cuh"
 #include "tc05.cuh"
@@ -17,18 +18,22 @@ namespace muse {
 
 typedef __nv_bfloat16 bf16;
 int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
+int make_tmap_bf16_nd(void* out_map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                      const uint32_t* box);
 
 namespace st {
 constexpr int D = 128, TI = 128, NU = 64, THREADS = 256;
 constexpr int kTile = TI * D * 2, kKeys = NU * D * 2, kW = TI * NU * 2;
 constexpr int oQhi = 0, oQlo = oQhi + kTile, oK = oQlo + kTile, oV = oK + kKeys, oWhi = oV + kKeys, oWlo = oWhi + kW;
-constexpr int total = oWlo + kW + 1024;
+constexpr int oStage = oWlo + kW;                 // three 32 KB snapshot tiles (kappa hi, kappa lo, nu) leaving by TMA
+constexpr int total = oStage + 3 * kTile + 1024;
 constexpr uint32_t cL = 0, cUk = 64, cUv = 192;
 }  // namespace st
 
 __global__ void __launch_bounds__(st::THREADS, 1)
 k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_constant__ CUtensorMap tm_V,
-               const int32_t* __restrict__ off_k, const float* __restrict__ qbar, SummPtrs sp, int* __restrict__ status) {
+               const __grid_constant__ CUtensorMap tm_okhi, const __grid_constant__ CUtensorMap tm_oklo,
+               const __grid_constant__ CUtensorMap tm_onu, const int32_t* __restrict__ off_k, const float* __restrict__ qbar, SummPtrs sp, int* __restrict__ status) {
   using namespace st;
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar_kv, bar1, bar2;
@@ -174,35 +179,39 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
       sp.mu[ent] = m_;
       sp.beta[ent] = some ? m_ - T * inv : -INFINITY;
     }
-    unsigned char* stage = sm + oWhi;                                 // 32 KB = [128 rows][256 B]
+    // kappa hi / lo (warpgroup 0) and nu (warpgroup 1) as swizzled [128 rows][2 x 128 B] tiles; they leave
+    // by TMA (rows of consecutive query clusters are Ck entries apart in memory) while the next plane is computed
+    if (tid == 0) tc::tma_store_wait_read();                           // the previous plane's stores have read the tiles
+    __syncthreads();
 #pragma unroll
-    for (int round = 0; round < 3; ++round) {                         // 0: kappa hi, 1: kappa lo, 2: nu
-      __syncthreads();
-      if ((round < 2 && wg == 0) || (round == 2 && wg == 1)) {
+    for (int ck = 0; ck < D / 8; ++ck) {
+      uint32_t w[4], wl_[4];
 #pragma unroll
-        for (int ck = 0; ck < D / 8; ++ck) {
-          uint32_t w[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const float x0 = acc[ck * 8 + 2 * e] * inv, x1 = acc[ck * 8 + 2 * e + 1] * inv;
-            __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
-            if (round == 1) hh = __floats2bfloat162_rn(x0 - __low2float(hh), x1 - __high2float(hh));
-            w[e] = *reinterpret_cast<uint32_t*>(&hh);
-          }
-          *reinterpret_cast<uint4*>(stage + row * 256 + ((ck ^ (row & 15)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-        }
+      for (int e = 0; e < 4; ++e) {
+        const float x0 = acc[ck * 8 + 2 * e] * inv, x1 = acc[ck * 8 + 2 * e + 1] * inv;
+        __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
+        __nv_bfloat162 ll = __floats2bfloat162_rn(x0 - __low2float(hh), x1 - __high2float(hh));
+        w[e] = *reinterpret_cast<uint32_t*>(&hh); wl_[e] = *reinterpret_cast<uint32_t*>(&ll);
       }
-      __syncthreads();
-      bf16* dst = (bf16*)(round == 0 ? sp.khi : round == 1 ? sp.klo : sp.nu);
-      for (int e = tid; e < TI * (D / 8); e += THREADS) {
-        const int r = e >> 4, ck = e & 15;
-        if (i0 + r < dm.Cq) {
-          const uint4 val = *reinterpret_cast<const uint4*>(stage + r * 256 + ((ck ^ (r & 15)) << 4));
-          *reinterpret_cast<uint4*>(dst + ((ent_row0 + i0 + r) * dm.Ck + j) * D + ck * 8) = val;
-        }
+      const uint32_t off = (ck >> 3) * TI * 128 + tc::sw128_off(row, ck & 7);
+      if (wg == 0) {
+        *reinterpret_cast<uint4*>(sm + oStage + off) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(sm + oStage + kTile + off) = make_uint4(wl_[0], wl_[1], wl_[2], wl_[3]);
+      } else {
+        *reinterpret_cast<uint4*>(sm + oStage + 2 * kTile + off) = make_uint4(w[0], w[1], w[2], w[3]);
       }
     }
+    tc::fence_async_smem();
+    __syncthreads();
+    if (tid == 0 && ok) {
+      const int P = pq * dm.SB + pl;
+      tc::tma_store_4d(&tm_okhi, sm + oStage, 0, j, i0, P);              tc::tma_store_4d(&tm_okhi, sm + oStage + TI * 128, 64, j, i0, P);
+      tc::tma_store_4d(&tm_oklo, sm + oStage + kTile, 0, j, i0, P);      tc::tma_store_4d(&tm_oklo, sm + oStage + kTile + TI * 128, 64, j, i0, P);
+      tc::tma_store_4d(&tm_onu, sm + oStage + 2 * kTile, 0, j, i0, P);   tc::tma_store_4d(&tm_onu, sm + oStage + 2 * kTile + TI * 128, 64, j, i0, P);
+      tc::tma_store_commit();
+    }
   }
+  if (tid == 0) tc::tma_store_wait_all();
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tbase, 512);
@@ -216,10 +225,18 @@ int summarize_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* o
   CUtensorMap tK, tV;
   int rc = make_tmap_bf16_rows(&tK, Kp, (uint64_t)d.B * d.Hkv * d.N, st::D, st::NU);
   if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tV, Vp, (uint64_t)d.B * d.Hkv * d.N, st::D, st::NU);
+  // outputs as 4-D tensors (d, j, i, head * planes + plane); a box is 128 query clusters of one key cluster
+  CUtensorMap okhi, oklo, onu;
+  const uint64_t dims[4] = {(uint64_t)st::D, (uint64_t)d.Ck, (uint64_t)d.Cq, (uint64_t)d.B * d.Hq * d.SB};
+  const uint64_t strides[3] = {(uint64_t)st::D * 2, (uint64_t)d.Ck * st::D * 2, (uint64_t)d.Cq * d.Ck * st::D * 2};
+  const uint32_t box[4] = {64, 1, (uint32_t)st::TI, 1};
+  if (rc == MUSE_OK) rc = make_tmap_bf16_nd(&okhi, sp.khi, 4, dims, strides, box);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_nd(&oklo, sp.klo, 4, dims, strides, box);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_nd(&onu, sp.nu, 4, dims, strides, box);
   if (rc != MUSE_OK) return rc;
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, st::total));
   prof_mark("k_summarize_tc", stream);
-  k_summarize_tc<<<dim3(d.Ck, cdiv(d.Cq, st::TI), d.B * d.Hq), st::THREADS, st::total, stream>>>(d, tK, tV, off_k, qbar, sp, status);
+  k_summarize_tc<<<dim3(d.Ck, cdiv(d.Cq, st::TI), d.B * d.Hq), st::THREADS, st::total, stream>>>(d, tK, tV, okhi, oklo, onu, off_k, qbar, sp, status);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }

@@ -49,4 +49,21 @@ int make_tmap_bf16_pitched(void* out_map, const void* base, uint64_t rows, uint6
   return r == CUDA_SUCCESS ? MUSE_OK : MUSE_ERR_CUDA;
 }
 
+// bf16 tensor of rank 3 or 4 (dims innermost first, strides in bytes for dims 1..rank-1, multiples
+// of 16), box given per dimension with 64 innermost elements, 128-byte swizzle.  Used for tiled
+// stores whose rows are not adjacent in memory (a box of 128 rows x 1 x 64 elements).
+int make_tmap_bf16_nd(void* out_map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                      const uint32_t* box) {
+  EncodeTiledFn fn = encode_fn();
+  if (fn == nullptr || rank < 3 || rank > 4) return MUSE_ERR_CUDA;
+  cuuint64_t gdim[4], gstride[3];
+  cuuint32_t bx[4], estr[4];
+  for (int k = 0; k < rank; ++k) { gdim[k] = dims[k]; bx[k] = box[k]; estr[k] = 1; }
+  for (int k = 0; k + 1 < rank; ++k) gstride[k] = strides_bytes[k];
+  CUresult r = fn(reinterpret_cast<CUtensorMap*>(out_map), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, (cuuint32_t)rank, const_cast<void*>(base),
+                  gdim, gstride, bx, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MUSE_OK : MUSE_ERR_CUDA;
+}
+
 }  // namespace muse
