@@ -77,20 +77,44 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
 #pragma unroll
   for (int d = 0; d < D; ++d) acc[d] = 0.f;
   float M = -INFINITY, s = 0.f, T = 0.f;           // running max, mass and sum of w * logit (all relative to M)
+#ifdef MUSE_PHASE_CLOCKS
+  long long pc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  long long t_ = clock64();
+#define PCLK(k) { long long n_ = clock64(); pc[k] += n_ - t_; t_ = n_; }
+#else
+#define PCLK(k)
+#endif
 
+  // The cluster's keys are contiguous in bucket order, so its chunks (at most 64 keys, never across a
+  // bucket boundary) form one sequence; thread 0 starts the load of chunk n + 1 as soon as the MMAs of
+  // chunk n have released the key / value tiles, so that it lands while the snapshot is written.
+  // A bucket usually holds far fewer than 64 keys: only the 16-key groups in use are loaded and contracted.
+  auto issue_kv = [&](int c0, int nk) {
+    const int ng_ = (nk + 15) >> 4;
+    tc::mbar_expect_tx(&bar_kv, ng_ * 4 * (16 * 128));
+    const int r = (int)((size_t)pk * dm.N + c0);
+    for (int g = 0; g < ng_; ++g) {
+      tc::tma_load_2d(sm + oK + g * 16 * 128, &tm_K, 0, r + 16 * g, &bar_kv); tc::tma_load_2d(sm + oK + NU * 128 + g * 16 * 128, &tm_K, 64, r + 16 * g, &bar_kv);
+      tc::tma_load_2d(sm + oV + g * 16 * 128, &tm_V, 0, r + 16 * g, &bar_kv); tc::tma_load_2d(sm + oV + NU * 128 + g * 16 * 128, &tm_V, 64, r + 16 * g, &bar_kv);
+    }
+  };
+  auto issue_after = [&](int c_end) {                  // the chunk that starts at key c_end, if any
+    int npl = 0;
+    while (npl < dm.SB && off[npl + 1] <= c_end) ++npl;
+    if (npl < dm.SB) issue_kv(c_end, min(NU, off[npl + 1] - c_end));
+  };
+  if (tid == 0) issue_after(off[0]);
   for (int pl = 0; pl < dm.SB && ok; ++pl) {
     const int p0 = off[pl], p1 = off[pl + 1];
     for (int c0 = p0; c0 < p1 && ok; c0 += NU) {
       const int nk = min(NU, p1 - c0);
+      PCLK(0)
       __syncthreads();
+      const int ng = (nk + 15) >> 4;
       if (tid == 0) {
-        tc::mbar_expect_tx(&bar_kv, 2 * kKeys);
-        const int r = (int)((size_t)pk * dm.N + c0);
-        tc::tma_load_2d(sm + oK, &tm_K, 0, r, &bar_kv); tc::tma_load_2d(sm + oK + NU * 128, &tm_K, 64, r, &bar_kv);
-        tc::tma_load_2d(sm + oV, &tm_V, 0, r, &bar_kv); tc::tma_load_2d(sm + oV + NU * 128, &tm_V, 64, r, &bar_kv);
         if (!tc::mbar_wait(&bar_kv, ph_kv)) ok = false;
         tc::fence_after_sync();
-        const uint32_t idesc = tc::idesc_bf16(TI, NU, 0, 0);
+        const uint32_t idesc = tc::idesc_bf16(TI, 16 * ng, 0, 0);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks)
           tc::mma_bf16_ss(tbase + cL, tc::smem_desc_sw128(aQhi + (ks / 4) * TI * 128 + (ks % 4) * 32, 16, 1024),
@@ -106,26 +130,25 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
       if (!tc::mbar_wait(&bar1, ph1)) ok = false;
       ph1 ^= 1;
       tc::fence_after_sync();
-      // two sweeps over the 64 logits in TMEM (max, then weights) keep the register footprint small
+      PCLK(1)
+      // two sweeps over the logits in TMEM (max, then weights) keep the register footprint small
       float cm = -INFINITY;
+      for (int g = 0; g < ng; ++g) {
+        float v[16];
+        tc::tmem_ld16(tlane + cL + 16 * g, v);
 #pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        float v[32];
-        tc::tmem_ld32(tlane + cL + 32 * hh, v);
-#pragma unroll
-        for (int u = 0; u < 32; ++u) if (32 * hh + u < nk) cm = fmaxf(cm, v[u]);
+        for (int u = 0; u < 16; ++u) if (16 * g + u < nk) cm = fmaxf(cm, v[u]);
       }
       const float Mn = fmaxf(M, cm);
       const float sc = __expf(M - Mn);                 // 0 on the first keys (M = -inf)
       float ws = 0.f, wl = 0.f;
+      for (int g = 0; g < ng; ++g) {
+        float v[16];
+        tc::tmem_ld16(tlane + cL + 16 * g, v);
+        uint32_t pk_[8];
 #pragma unroll
-      for (int hh = 0; hh < 2; ++hh) {
-        float v[32];
-        tc::tmem_ld32(tlane + cL + 32 * hh, v);
-        uint32_t pk_[16];
-#pragma unroll
-        for (int u = 0; u < 32; u += 2) {
-          const bool in0 = 32 * hh + u < nk, in1 = 32 * hh + u + 1 < nk;
+        for (int u = 0; u < 16; u += 2) {
+          const bool in0 = 16 * g + u < nk, in1 = 16 * g + u + 1 < nk;
           const float w0 = in0 ? __expf(v[u] - Mn) : 0.f, w1 = in1 ? __expf(v[u + 1] - Mn) : 0.f;
           ws += w0 + w1;
           wl += (in0 ? w0 * v[u] : 0.f) + (in1 ? w1 * v[u + 1] : 0.f);
@@ -134,23 +157,22 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
           pk_[u >> 1] = wg == 0 ? *reinterpret_cast<uint32_t*>(&hb) : *reinterpret_cast<uint32_t*>(&lb);
         }
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch)
-          *reinterpret_cast<uint4*>(sm + (wg == 0 ? oWhi : oWlo) + tc::sw128_off(row, 4 * hh + ch)) = make_uint4(pk_[4 * ch], pk_[4 * ch + 1], pk_[4 * ch + 2], pk_[4 * ch + 3]);
+        for (int ch = 0; ch < 2; ++ch)
+          *reinterpret_cast<uint4*>(sm + (wg == 0 ? oWhi : oWlo) + tc::sw128_off(row, 2 * g + ch)) = make_uint4(pk_[4 * ch], pk_[4 * ch + 1], pk_[4 * ch + 2], pk_[4 * ch + 3]);
       }
       s = s * sc + ws; T = T * sc + wl; M = Mn;
       tc::fence_async_smem();
       tc::fence_before_sync();
       __syncthreads();
+      PCLK(2)
       if (tid == 0) {
         tc::fence_after_sync();
         const uint32_t idesc = tc::idesc_bf16(TI, D, 0, 1);          // A = W (K-major over keys), B = key rows (MN-major)
-#pragma unroll
-        for (int ks = 0; ks < NU / 16; ++ks) {
+        for (int ks = 0; ks < ng; ++ks) {
           tc::mma_bf16_ss(tbase + cUk, tc::smem_desc_sw128(aWhi + ks * 32, 16, 1024), tc::smem_desc_sw128(aK + ks * 16 * 128, NU * 128, 1024), idesc, ks > 0);
           tc::mma_bf16_ss(tbase + cUv, tc::smem_desc_sw128(aWhi + ks * 32, 16, 1024), tc::smem_desc_sw128(aV + ks * 16 * 128, NU * 128, 1024), idesc, ks > 0);
         }
-#pragma unroll
-        for (int ks = 0; ks < NU / 16; ++ks) {
+        for (int ks = 0; ks < ng; ++ks) {
           tc::mma_bf16_ss(tbase + cUk, tc::smem_desc_sw128(aWlo + ks * 32, 16, 1024), tc::smem_desc_sw128(aK + ks * 16 * 128, NU * 128, 1024), idesc, 1);
           tc::mma_bf16_ss(tbase + cUv, tc::smem_desc_sw128(aWlo + ks * 32, 16, 1024), tc::smem_desc_sw128(aV + ks * 16 * 128, NU * 128, 1024), idesc, 1);
         }
@@ -160,6 +182,8 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
       if (!tc::mbar_wait(&bar2, ph2)) ok = false;
       ph2 ^= 1;
       tc::fence_after_sync();
+      if (tid == 0 && ok) issue_after(c0 + nk);          // key / value tiles are free again
+      PCLK(3)
 #pragma unroll
       for (int d0 = 0; d0 < D; d0 += 32) {
         float v[32];
@@ -168,6 +192,10 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
         for (int e = 0; e < 32; ++e) acc[d0 + e] = fmaf(acc[d0 + e], sc, v[e]);
       }
       tc::fence_before_sync();
+      PCLK(4)
+#ifdef MUSE_PHASE_CLOCKS
+      pc[7] += 1;
+#endif
     }
     // ---- snapshot of plane pl: three 128 x 256-byte row tiles (kappa hi, kappa lo, nu) staged in the W region
     const bool some = s > 0.f;
@@ -210,7 +238,11 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
       tc::tma_store_4d(&tm_onu, sm + oStage + 2 * kTile, 0, j, i0, P);   tc::tma_store_4d(&tm_onu, sm + oStage + 2 * kTile + TI * 128, 64, j, i0, P);
       tc::tma_store_commit();
     }
+    PCLK(5)
   }
+#ifdef MUSE_PHASE_CLOCKS
+  if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 0 && blockIdx.z == 0) for (int k = 0; k < 8; ++k) status[56 + k] = (int)pc[k];
+#endif
   if (tid == 0) tc::tma_store_wait_all();
   tc::fence_before_sync();
   __syncthreads();
@@ -223,8 +255,8 @@ bool summarize_tc_supported(const Dims& d, int dtype) { return dtype == MUSE_BF1
 int summarize_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const float* qbar, const SummPtrs& sp,
                  int* status, cudaStream_t stream) {
   CUtensorMap tK, tV;
-  int rc = make_tmap_bf16_rows(&tK, Kp, (uint64_t)d.B * d.Hkv * d.N, st::D, st::NU);
-  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tV, Vp, (uint64_t)d.B * d.Hkv * d.N, st::D, st::NU);
+  int rc = make_tmap_bf16_rows(&tK, Kp, (uint64_t)d.B * d.Hkv * d.N, st::D, 16);       // boxes of 16 keys
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tV, Vp, (uint64_t)d.B * d.Hkv * d.N, st::D, 16);
   // outputs as 4-D tensors (d, j, i, head * planes + plane); a box is 128 query clusters of one key cluster
   CUtensorMap okhi, oklo, onu;
   const uint64_t dims[4] = {(uint64_t)st::D, (uint64_t)d.Ck, (uint64_t)d.Cq, (uint64_t)d.B * d.Hq * d.SB};
