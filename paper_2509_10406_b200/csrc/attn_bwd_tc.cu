@@ -11,6 +11,8 @@
 #include "common.cuh"
 #include "tc05.cuh"
 
+#include <cstdlib>
+
 namespace muse {
 
 typedef __nv_bfloat16 bf16;
@@ -580,6 +582,232 @@ k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
   bwd_teardown(c, SM::cols, tid, status);
 }
 
+// ================================================================================================
+// Fused retrieval backward (D = 128): one CTA per (key cluster j, head) walks every plane's group
+// of retrieving (query, slot) pairs in tiles of 128 pairs (pairs on the MMA M side), against the
+// cluster's keys in chunks of 64 (at most two chunks resident; longer clusters take another
+// sweep).  Per tile and key chunk:
+//   S = Q K^T, dP = dO V^T  ->  P = exp(sigma S - L), G = P (dP - delta)   (one thread per pair row)
+//   dQ   += G K                     [pairs][D]   written per pair as a bf16 row
+//   dV^T += dO^T P,  dK^T += Q^T G  [D][keys]    accumulated in TMEM over all tiles and planes
+// Q and dO rows are gathered once for all three products, one tile ahead (registers), their pair
+// ids two tiles ahead, across plane boundaries.  The CTA owns the cluster's keys for its head, so
+// dK and dV leave with plain coalesced read-modify-writes (thread = output dim).
+// ================================================================================================
+constexpr int kFusedThreads = 256, kFusedChunks = 2;
+
+struct FusedSmem {
+  static constexpr int D = 128;
+  static constexpr int q = 0, dO = q + kBM * D * 2, k = dO + kBM * D * 2, v = k + kFusedChunks * kBN * D * 2,
+                       p = v + kFusedChunks * kBN * D * 2, g = p + kBM * kBN * 2, total = g + kBM * kBN * 2 + 1024;
+  static constexpr uint32_t cS = 0, cDP = 64, cDQ = 128, cDV = 256, cDK = 384, cols = 512;
+};
+
+__global__ void __launch_bounds__(kFusedThreads, 1)
+k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO, const bf16* __restrict__ Kp,
+                   const bf16* __restrict__ Vp, const float* __restrict__ LSE, const float* __restrict__ delta,
+                   const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
+                   bf16* __restrict__ dq_part, float* __restrict__ dK_perm, float* __restrict__ dV_perm, int* __restrict__ status) {
+  typedef FusedSmem SM;
+  constexpr int D = SM::D, KC = kFusedChunks * kBN;        // keys per sweep
+  extern __shared__ __align__(1024) unsigned char sm_raw[];
+  __shared__ uint64_t bar[2];
+  __shared__ uint32_t tbase_s;
+  __shared__ int32_t pid_s[2][kBM];
+  const int tid = threadIdx.x, warp = tid >> 5, row = tid & 127, wg = tid >> 7;
+  const int j = blockIdx.x, pq = blockIdx.y;
+  const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
+  const int nkeys = dm.SB * dm.Ck;
+  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + j;                // group of plane pl: go[pl * Ck], go[pl * Ck + 1]
+  const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
+  const int k0 = ok[0], kall = ok[dm.SB];
+  // any retrieving pair at all?
+  bool any_pair = false;
+  for (int pl = 0; pl < dm.SB; ++pl) any_pair |= go[(size_t)pl * dm.Ck + 1] > go[(size_t)pl * dm.Ck];
+  if (!any_pair) return;
+  BwdCtx c;
+  bwd_setup(c, sm_raw, bar, &tbase_s, SM::cols, tid);
+  const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
+  const bf16* Kb = Kp + (size_t)pk * dm.N * D; const bf16* Vb = Vp + (size_t)pk * dm.N * D;
+  const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
+  const uint32_t qa = tc::smem_u32(c.sm + SM::q), da = tc::smem_u32(c.sm + SM::dO), ka = tc::smem_u32(c.sm + SM::k),
+                 va = tc::smem_u32(c.sm + SM::v), pa = tc::smem_u32(c.sm + SM::p), ga = tc::smem_u32(c.sm + SM::g);
+  const uint32_t tl = c.tbase + ((uint32_t)((warp & 3) * 32) << 16);
+  const float scale2 = dm.sigma * kLog2e;
+
+  // work items: (plane, first pair of the tile); a plane takes part in a sweep if it has pairs and, from the
+  // second sweep on, if it sees keys of that sweep
+  struct Item { int pl, t0, g1; };
+  for (int kc0 = k0; (kc0 < kall || kc0 == k0) && c.ok; kc0 += KC) {
+    const bool first_sweep = kc0 == k0;
+    auto plane_active = [&](int pl) {
+      const int g0 = go[(size_t)pl * dm.Ck], g1 = go[(size_t)pl * dm.Ck + 1];
+      return g1 > g0 && (first_sweep || ok[pl + 1] > kc0);
+    };
+    auto first_from = [&](int pl) {
+      Item it; it.pl = pl;
+      while (it.pl < dm.SB && !plane_active(it.pl)) ++it.pl;
+      if (it.pl < dm.SB) { it.t0 = go[(size_t)it.pl * dm.Ck]; it.g1 = go[(size_t)it.pl * dm.Ck + 1]; } else { it.t0 = 0; it.g1 = 0; }
+      return it;
+    };
+    auto next_of = [&](const Item& a) {
+      if (a.pl >= dm.SB) return a;
+      if (a.t0 + kBM < a.g1) { Item it = a; it.t0 += kBM; return it; }
+      return first_from(a.pl + 1);
+    };
+    // key / value chunks of this sweep
+    __syncthreads();
+    const int nkc = min(KC, kall - kc0);                    // keys of the sweep that any plane sees
+#pragma unroll
+    for (int ch = 0; ch < kFusedChunks; ++ch) {
+      const int n = min(kBN, max(0, nkc - ch * kBN));
+      fill_tile<D, kBN, kFusedThreads>(c.sm + SM::k + ch * kBN * D * 2, n, [&](int r) { return Kb + (size_t)(kc0 + ch * kBN + r) * D; }, tid);
+      fill_tile<D, kBN, kFusedThreads>(c.sm + SM::v + ch * kBN * D * 2, n, [&](int r) { return Vb + (size_t)(kc0 + ch * kBN + r) * D; }, tid);
+    }
+    bool started[kFusedChunks] = {false, false};            // dV^T / dK^T of chunk ch hold something
+
+    TileRegs<D, kBM, kFusedThreads> qreg, oreg;
+    float Lreg = 0.f, dreg = 0.f;
+    int pidreg = 0;
+    auto load_pids = [&](const Item& it) {
+      if (tid < kBM) pidreg = (it.pl < dm.SB && it.t0 + tid < it.g1) ? __ldg(pr + it.t0 + tid) : 0;
+    };
+    auto load_rows = [&](const Item& it, const int32_t* pid) {
+      const int nq = min(kBM, it.g1 - it.t0);
+      tile_ldg<D, kBM, kFusedThreads>(qreg, nq, [&](int r) { return Qb + (size_t)(pid[r] / dm.m) * D; }, tid);
+      tile_ldg<D, kBM, kFusedThreads>(oreg, nq, [&](int r) { return dOb + (size_t)(pid[r] / dm.m) * D; }, tid);
+      const size_t tt = (size_t)pq * dm.N + pid[row] / dm.m;
+      Lreg = row < nq ? LSE[tt] * kLog2e : 0.f;
+      dreg = row < nq ? delta[tt] : 0.f;
+    };
+    Item cur = first_from(0), nxt = next_of(cur), nn = next_of(nxt);
+    load_pids(cur);
+    if (tid < kBM) pid_s[0][tid] = pidreg;
+    load_pids(nxt);
+    __syncthreads();
+    if (cur.pl < dm.SB) load_rows(cur, pid_s[0]);
+    int buf = 0;
+    while (cur.pl < dm.SB && c.ok) {
+      const int nq = min(kBM, cur.g1 - cur.t0);
+      const int vis = min(KC, max(0, ok[cur.pl + 1] - kc0));            // keys of this sweep that the plane sees
+      const int nch = (vis + kBN - 1) / kBN;
+      tile_sts<D, kBM, kFusedThreads>(qreg, c.sm + SM::q, tid);
+      tile_sts<D, kBM, kFusedThreads>(oreg, c.sm + SM::dO, tid);
+      if (tid < kBM) pid_s[buf ^ 1][tid] = pidreg;                      // pair ids of the next tile
+      const float L2 = Lreg, dl = dreg;
+      const int my_pid = pid_s[buf][row];
+      tc::fence_async_smem();
+      tc::fence_before_sync();
+      __syncthreads();                                                  // tiles and pid_s[buf ^ 1] visible
+      if (nxt.pl < dm.SB) load_rows(nxt, pid_s[buf ^ 1]);               // gathers fly while this tile is processed
+      load_pids(nn);
+      for (int ch = 0; ch < nch && c.ok; ++ch) {
+        const uint32_t kac = ka + ch * kBN * D * 2, vac = va + ch * kBN * D * 2;
+        if (tid == 0) {
+          tc::fence_after_sync();
+          const uint32_t idesc = tc::idesc_bf16(kBM, kBN, 0, 0);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase + SM::cS, desc_k<kBM>(qa, ks), desc_k<kBN>(kac, ks), idesc, ks > 0);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase + SM::cDP, desc_k<kBM>(da, ks), desc_k<kBN>(vac, ks), idesc, ks > 0);
+          tc::mma_commit(&c.bar[0]);
+        }
+        __syncwarp();
+        if (!tc::mbar_wait(&c.bar[0], c.ph0)) { c.ok = false; break; }
+        c.ph0 ^= 1;
+        tc::fence_after_sync();
+        {
+          const int visc = min(kBN, vis - ch * kBN);
+          float sv[32], dp[32], pv[32], gv[32];
+          tc::tmem_ld32(tl + SM::cS + 32 * wg, sv);
+          tc::tmem_ld32(tl + SM::cDP + 32 * wg, dp);
+#pragma unroll
+          for (int i = 0; i < 32; ++i) {
+            const float e = tc::fast_exp2(sv[i] * scale2 - L2);
+            pv[i] = (row < nq && 32 * wg + i < visc) ? e : 0.f;
+            gv[i] = pv[i] * (dp[i] - dl);
+          }
+          store_row32(c.sm + SM::p, row, wg, pv);
+          store_row32(c.sm + SM::g, row, wg, gv);
+        }
+        tc::fence_async_smem();
+        tc::fence_before_sync();
+        __syncthreads();
+        if (tid == 0) {
+          tc::fence_after_sync();
+          const uint32_t id_dq = tc::idesc_bf16(kBM, D, 0, 1);          // A = G (contraction over keys), B = key rows MN-major
+          const uint32_t id_t = tc::idesc_bf16(D, kBN, 1, 1);           // A = dO / Q tile and B = P / G tile, both contracted over pairs
+#pragma unroll
+          for (int ks = 0; ks < kBN / 16; ++ks)
+            tc::mma_bf16_ss(c.tbase + SM::cDQ, tc::smem_desc_sw128(ga + ks * 32, 16, 1024), desc_mn<kBN>(kac, ks), id_dq, ch > 0 || ks > 0);
+#pragma unroll
+          for (int ks = 0; ks < kBM / 16; ++ks)
+            tc::mma_bf16_ss(c.tbase + SM::cDV + ch * kBN, desc_mn<kBM>(da, ks), tc::smem_desc_sw128(pa + ks * 16 * 128, kBM * 128, 1024), id_t,
+                            started[ch] || ks > 0);
+#pragma unroll
+          for (int ks = 0; ks < kBM / 16; ++ks)
+            tc::mma_bf16_ss(c.tbase + SM::cDK + ch * kBN, desc_mn<kBM>(qa, ks), tc::smem_desc_sw128(ga + ks * 16 * 128, kBM * 128, 1024), id_t,
+                            started[ch] || ks > 0);
+          tc::mma_commit(&c.bar[1]);
+        }
+        started[ch] = true;
+        __syncwarp();
+        if (!tc::mbar_wait(&c.bar[1], c.ph1)) { c.ok = false; break; }
+        c.ph1 ^= 1;
+        tc::fence_after_sync();
+      }
+      if (c.ok) {
+        // bf16 dQ row per (query, slot); each warpgroup converts and stores half of it.  Later sweeps add to it.
+        bf16* dst = dq_part + ((size_t)pq * dm.N * dm.m + my_pid) * D + wg * (D / 2);
+        const uint32_t tq = tl + SM::cDQ + wg * (D / 2);
+#pragma unroll
+        for (int d0 = 0; d0 < D / 2; d0 += 32) {
+          float v[32];
+          if (nch > 0) tc::tmem_ld32(tq + d0, v);
+          if (row < nq) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 8) {
+              float x[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) x[e] = nch > 0 ? v[i + e] * dm.sigma : 0.f;
+              if (!first_sweep) {
+                const float4 o0 = ld4(dst + d0 + i), o1 = ld4(dst + d0 + i + 4);
+                x[0] += o0.x; x[1] += o0.y; x[2] += o0.z; x[3] += o0.w; x[4] += o1.x; x[5] += o1.y; x[6] += o1.z; x[7] += o1.w;
+              }
+              uint32_t w[4];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) { __nv_bfloat162 b2 = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]); w[e] = *reinterpret_cast<uint32_t*>(&b2); }
+              *reinterpret_cast<uint4*>(dst + d0 + i) = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          }
+        }
+      }
+      tc::fence_before_sync();
+      cur = nxt; nxt = nn; nn = next_of(nn); buf ^= 1;
+    }
+    // dV (warpgroup 0) and dK (warpgroup 1) of this sweep's keys: thread = output dim, one key per column
+#pragma unroll
+    for (int ch = 0; ch < kFusedChunks; ++ch) {
+      if (!started[ch]) continue;                                       // uniform over the CTA
+      const int n = min(kBN, nkc - ch * kBN);
+      float* dst = (wg == 0 ? dV_perm : dK_perm) + ((size_t)pq * dm.N + kc0 + ch * kBN) * D + row;
+      const float f = wg == 0 ? 1.f : dm.sigma;
+#pragma unroll
+      for (int u0 = 0; u0 < kBN; u0 += 32) {
+        float v[32];
+        tc::tmem_ld32(tl + (wg == 0 ? SM::cDV : SM::cDK) + ch * kBN + u0, v);
+        if (c.ok) {
+#pragma unroll
+          for (int u = 0; u < 32; ++u)
+            if (u0 + u < n) dst[(size_t)(u0 + u) * D] += v[u] * f;
+        }
+      }
+    }
+    tc::fence_before_sync();
+  }
+  bwd_teardown(c, SM::cols, tid, status);
+}
+
 // ---- launchers ------------------------------------------------------------------------------------
 #define MUSE_TC_LAUNCH(KERNEL, SMEM, NT, GRID, ...)                                                                  \
   do {                                                                                                            \
@@ -610,6 +838,14 @@ int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, con
                const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, void* dq_part,
                float* dK_perm, float* dV_perm, int* status, cudaStream_t st) {
   const int pq = d.B * d.Hq;
+  if (d.D == 128 && getenv("MUSE_RET_BWD_SPLIT") == nullptr) {
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_bwd_fused_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, FusedSmem::total));
+    prof_mark("k_ret_bwd_fused_tc", st);
+    k_ret_bwd_fused_tc<<<dim3(d.Ck, pq), kFusedThreads, FusedSmem::total, st>>>(d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp, (const bf16*)Vp,
+                                                                               LSE, delta, off_k, goff, pairs, (bf16*)dq_part, dK_perm, dV_perm, status);
+    MUSE_LAUNCH_OK();
+    return MUSE_OK;
+  }
   prof_mark("k_ret_bwd_dkdv_tc", st);
   MUSE_TC_LAUNCH(k_ret_bwd_dkdv_tc, KeysSmem, kKeysThreads, dim3(d.Ck, d.SB * kRetSplit, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
                  (const bf16*)Vp, LSE, delta, off_k, goff, pairs, dK_perm, dV_perm, status);

@@ -15,6 +15,8 @@ namespace muse {
 
 typedef __nv_bfloat16 bf16;
 int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
+int make_tmap_bf16_nd(void* out_map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                      const uint32_t* box);
 
 namespace fb {
 constexpr int D = 128, TJ = 128, NR = 64, NP = 2, THREADS = 256;
@@ -36,7 +38,8 @@ __device__ __forceinline__ float fast_exp2(float x) {
 
 __global__ void __launch_bounds__(fb::THREADS, 1)
 k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_constant__ CUtensorMap tm_klo,
-             const __grid_constant__ CUtensorMap tm_nu, const bf16* __restrict__ Q, const bf16* __restrict__ dO,
+             const __grid_constant__ CUtensorMap tm_nu, const __grid_constant__ CUtensorMap tm_gka,
+             const __grid_constant__ CUtensorMap tm_gnu, const bf16* __restrict__ Q, const bf16* __restrict__ dO,
              const float* __restrict__ qbar, const float* __restrict__ LSE, const float* __restrict__ delta,
              const int32_t* __restrict__ off_q, const int32_t* __restrict__ perm_q, const int32_t* __restrict__ sel,
              const float* __restrict__ beta, float* __restrict__ dQacc, bf16* __restrict__ dkappa,
@@ -111,6 +114,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       long long k0_ = clock64(), k1_ = 0, k2_ = 0, k3_ = 0, k4_ = 0;
 #endif
       if (tid == 0) {
+        tc::tma_store_wait_read();            // the previous tile's gradient stores have read the kappa_hi / nu buffers
         tc::mbar_expect_tx(&bar_full, 3 * kTile);
         const int row = (int)(ent0 + (size_t)jt * TJ);
         tc::tma_load_2d(sm + oHi, &tm_khi, 0, row, &bar_full); tc::tma_load_2d(sm + oHi + TJ * 128, &tm_khi, 64, row, &bar_full);
@@ -284,18 +288,18 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       }
       (void)dst;
       dots[wg][L] = dot;
+      // the two gradient tiles leave by TMA: 128 rows of 256 bytes each, Cq entries apart in the
+      // [plane][j][i] layout (adjacent in the [plane][i][j] one)
+      tc::fence_async_smem();
       __syncthreads();
-      if (ok) {
-        for (int e = tid; e < 2 * TJ * (D / 8); e += THREADS) {
-          const int arr = e / (TJ * (D / 8)), r = (e / (D / 8)) % TJ, ch = e % (D / 8);
-          const size_t ge = grad_by_key_cluster ? (((size_t)pq * dm.SB + pl) * Ck + jt * TJ + r) * dm.Cq + i : ent0 + (size_t)jt * TJ + r;
-          const uint4 val = *reinterpret_cast<const uint4*>(sm + (arr == 0 ? oNu : oHi) + (ch >> 3) * TJ * 128 + tc::sw128_off(r, ch & 7));
-          *reinterpret_cast<uint4*>((arr == 0 ? dnu : dkappa) + ge * D + ch * 8) = val;
-        }
+      if (tid == 0 && ok) {
+        const int c1 = grad_by_key_cluster ? i : 0;
+        const int c2 = grad_by_key_cluster ? (pq * dm.SB + pl) * Ck + jt * TJ : (int)(ent0 + (size_t)jt * TJ);
+        tc::tma_store_3d(&tm_gnu, sm + oNu, 0, c1, c2); tc::tma_store_3d(&tm_gnu, sm + oNu + TJ * 128, 64, c1, c2);
+        tc::tma_store_3d(&tm_gka, sm + oHi, 0, c1, c2); tc::tma_store_3d(&tm_gka, sm + oHi + TJ * 128, 64, c1, c2);
+        tc::tma_store_commit();
       }
-      tc::fence_async_smem();          // generic accesses to the tiles are ordered before the next TMA writes
       tc::fence_before_sync();
-      __syncthreads();
       if (wg == 0 && ok) dS[gent] = gtot - dots[0][L] - dots[1][L];
 #ifdef MUSE_PHASE_CLOCKS
       k4_ = clock64();
@@ -325,6 +329,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   }
   tc::fence_before_sync();
   __syncthreads();
+  if (tid == 0) tc::tma_store_wait_all();
   if (warp == 0) tc::tmem_dealloc(tbase, 512);
   if (!ok && tid == 0) atomicExch(status, 4);
 }
@@ -341,12 +346,21 @@ int far_bwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const void* dO,
   int rc = make_tmap_bf16_rows(&khi, sp.khi, ent, fb::D, fb::TJ);
   if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&klo, sp.klo, ent, fb::D, fb::TJ);
   if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&nu, sp.nu, ent, fb::D, fb::TJ);
+  // gradient tensors for the tiled stores: (d, i, plane * Ck + j) when grouped by key cluster, else (d, 1, entry)
+  CUtensorMap gka, gnu;
+  const uint64_t rows_j = (uint64_t)d.B * d.Hq * d.SB * d.Ck;
+  const uint64_t dims_a[3] = {(uint64_t)fb::D, (uint64_t)d.Cq, rows_j}, str_a[2] = {(uint64_t)fb::D * 2, (uint64_t)d.Cq * fb::D * 2};
+  const uint64_t dims_b[3] = {(uint64_t)fb::D, 1, ent}, str_b[2] = {(uint64_t)fb::D * 2, (uint64_t)fb::D * 2};
+  const uint32_t box[3] = {64, 1, (uint32_t)fb::TJ};
+  if (rc == MUSE_OK) rc = make_tmap_bf16_nd(&gka, dkappa, 3, grad_by_key_cluster ? dims_a : dims_b, grad_by_key_cluster ? str_a : str_b, box);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_nd(&gnu, dnu, 3, grad_by_key_cluster ? dims_a : dims_b, grad_by_key_cluster ? str_a : str_b, box);
   if (rc != MUSE_OK) return rc;
+  if (ent >= (1ull << 31)) return MUSE_ERR_UNSUPPORTED;      // 32-bit tile coordinates
   const size_t smem = (size_t)fb::oMask + (size_t)fb::NP * fb::NR * (d.Ck / 32) * 4 + 1024;
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_bwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prof_mark("k_far_bwd_tc", st);
   k_far_bwd_tc<<<dim3(d.Cq, d.SB, d.B * d.Hq), fb::THREADS, smem, st>>>(
-      d, khi, klo, nu, (const bf16*)Q, (const bf16*)dO, qbar, LSE, delta, off_q, perm_q, sel, sp.beta, dQacc, (bf16*)dkappa,
+      d, khi, klo, nu, gka, gnu, (const bf16*)Q, (const bf16*)dO, qbar, LSE, delta, off_q, perm_q, sel, sp.beta, dQacc, (bf16*)dkappa,
       (bf16*)dnu, dS, grad_by_key_cluster, status);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
