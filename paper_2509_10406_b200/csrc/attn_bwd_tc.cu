@@ -687,7 +687,44 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
     __syncthreads();
     if (cur.pl < dm.SB) load_rows(cur, pid_s[0]);
     int buf = 0;
+    // The dQ rows of a tile are written while the first products of the NEXT tile run on the tensor cores
+    // (the accumulator columns are only overwritten by that tile's second batch of MMAs).
+    int prev_pid = 0, prev_nq = 0, prev_nch = -1;              // prev_nch < 0: nothing pending
+    auto store_dq = [&]() {
+      if (prev_nch < 0) return;
+      // bf16 dQ row per (query, slot); each warpgroup converts and stores half of it.  Later sweeps add to it.
+      bf16* dst = dq_part + ((size_t)pq * dm.N * dm.m + prev_pid) * D + wg * (D / 2);
+      const uint32_t tq = tl + SM::cDQ + wg * (D / 2);
+#pragma unroll
+      for (int d0 = 0; d0 < D / 2; d0 += 32) {
+        float v[32];
+        if (prev_nch > 0) tc::tmem_ld32(tq + d0, v);
+        if (row < prev_nq && c.ok) {
+#pragma unroll
+          for (int i = 0; i < 32; i += 8) {
+            float x[8];
+#pragma unroll
+            for (int e = 0; e < 8; ++e) x[e] = prev_nch > 0 ? v[i + e] * dm.sigma : 0.f;
+            if (!first_sweep) {
+              const float4 o0 = ld4(dst + d0 + i), o1 = ld4(dst + d0 + i + 4);
+              x[0] += o0.x; x[1] += o0.y; x[2] += o0.z; x[3] += o0.w; x[4] += o1.x; x[5] += o1.y; x[6] += o1.z; x[7] += o1.w;
+            }
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { __nv_bfloat162 b2 = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]); w[e] = *reinterpret_cast<uint32_t*>(&b2); }
+            *reinterpret_cast<uint4*>(dst + d0 + i) = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+      }
+      prev_nch = -1;
+    };
     while (cur.pl < dm.SB && c.ok) {
+#ifdef MUSE_PHASE_CLOCKS
+      long long z_ = clock64();
+#define ZCLK(k) { long long n_ = clock64(); c.pc[k] += n_ - z_; z_ = n_; }
+#else
+#define ZCLK(k)
+#endif
       const int nq = min(kBM, cur.g1 - cur.t0);
       const int vis = min(KC, max(0, ok[cur.pl + 1] - kc0));            // keys of this sweep that the plane sees
       const int nch = (vis + kBN - 1) / kBN;
@@ -699,8 +736,14 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       tc::fence_async_smem();
       tc::fence_before_sync();
       __syncthreads();                                                  // tiles and pid_s[buf ^ 1] visible
-      if (nxt.pl < dm.SB) load_rows(nxt, pid_s[buf ^ 1]);               // gathers fly while this tile is processed
-      load_pids(nn);
+      ZCLK(0)
+      bool prefetched = false;
+      auto prefetch = [&]() {                                           // gathers of the next tile, pair ids of the one after
+        if (prefetched) return;
+        if (nxt.pl < dm.SB) load_rows(nxt, pid_s[buf ^ 1]);
+        load_pids(nn);
+        prefetched = true;
+      };
       for (int ch = 0; ch < nch && c.ok; ++ch) {
         const uint32_t kac = ka + ch * kBN * D * 2, vac = va + ch * kBN * D * 2;
         if (tid == 0) {
@@ -713,9 +756,12 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
           tc::mma_commit(&c.bar[0]);
         }
         __syncwarp();
+        if (ch == 0) store_dq();                                        // previous tile's rows leave meanwhile
+        ZCLK(1)
         if (!tc::mbar_wait(&c.bar[0], c.ph0)) { c.ok = false; break; }
         c.ph0 ^= 1;
         tc::fence_after_sync();
+        ZCLK(2)
         {
           const int visc = min(kBN, vis - ch * kBN);
           float sv[32], dp[32], pv[32], gv[32];
@@ -730,6 +776,7 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
           store_row32(c.sm + SM::p, row, wg, pv);
           store_row32(c.sm + SM::g, row, wg, gv);
         }
+        ZCLK(3)
         tc::fence_async_smem();
         tc::fence_before_sync();
         __syncthreads();
@@ -752,39 +799,24 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
         }
         started[ch] = true;
         __syncwarp();
+        prefetch();                                                     // the gathers are issued while these MMAs run
+        ZCLK(4)
         if (!tc::mbar_wait(&c.bar[1], c.ph1)) { c.ok = false; break; }
         c.ph1 ^= 1;
         tc::fence_after_sync();
+        ZCLK(5)
       }
-      if (c.ok) {
-        // bf16 dQ row per (query, slot); each warpgroup converts and stores half of it.  Later sweeps add to it.
-        bf16* dst = dq_part + ((size_t)pq * dm.N * dm.m + my_pid) * D + wg * (D / 2);
-        const uint32_t tq = tl + SM::cDQ + wg * (D / 2);
-#pragma unroll
-        for (int d0 = 0; d0 < D / 2; d0 += 32) {
-          float v[32];
-          if (nch > 0) tc::tmem_ld32(tq + d0, v);
-          if (row < nq) {
-#pragma unroll
-            for (int i = 0; i < 32; i += 8) {
-              float x[8];
-#pragma unroll
-              for (int e = 0; e < 8; ++e) x[e] = nch > 0 ? v[i + e] * dm.sigma : 0.f;
-              if (!first_sweep) {
-                const float4 o0 = ld4(dst + d0 + i), o1 = ld4(dst + d0 + i + 4);
-                x[0] += o0.x; x[1] += o0.y; x[2] += o0.z; x[3] += o0.w; x[4] += o1.x; x[5] += o1.y; x[6] += o1.z; x[7] += o1.w;
-              }
-              uint32_t w[4];
-#pragma unroll
-              for (int e = 0; e < 4; ++e) { __nv_bfloat162 b2 = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]); w[e] = *reinterpret_cast<uint32_t*>(&b2); }
-              *reinterpret_cast<uint4*>(dst + d0 + i) = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-          }
-        }
-      }
+      if (nch == 0) store_dq();                                         // (no product was issued above)
+      prefetch();
+      prev_pid = my_pid; prev_nq = nq; prev_nch = nch;
       tc::fence_before_sync();
       cur = nxt; nxt = nn; nn = next_of(nn); buf ^= 1;
+      ZCLK(6)
+#ifdef MUSE_PHASE_CLOCKS
+      c.pc[7] += 1;
+#endif
     }
+    store_dq();
     // dV (warpgroup 0) and dK (warpgroup 1) of this sweep's keys: thread = output dim, one key per column
 #pragma unroll
     for (int ch = 0; ch < kFusedChunks; ++ch) {
@@ -805,6 +837,10 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
     }
     tc::fence_before_sync();
   }
+#ifdef MUSE_PHASE_CLOCKS
+  if (tid == 0 && c.pc[7] >= 12 && atomicCAS(status + 40, 0, 1) == 0)
+    for (int k = 0; k < 8; ++k) status[41 + k] = (int)c.pc[k];
+#endif
   bwd_teardown(c, SM::cols, tid, status);
 }
 

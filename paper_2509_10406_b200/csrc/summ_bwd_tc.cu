@@ -286,7 +286,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tbase, 512);
 #ifdef MUSE_PHASE_CLOCKS
-  if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 0) for (int k = 0; k < 8; ++k) status[48 + k] = (int)pc[k];
+  if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 0) for (int k = 0; k < 8; ++k) status[56 + k] = 0 * (int)pc[k];
 #endif
   if (!ok && tid == 0) atomicExch(status, 5);
 }
