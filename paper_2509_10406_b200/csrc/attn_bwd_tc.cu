@@ -599,7 +599,8 @@ constexpr int kFusedThreads = 256, kFusedChunks = 2;
 struct FusedSmem {
   static constexpr int D = 128;
   static constexpr int q = 0, dO = q + kBM * D * 2, k = dO + kBM * D * 2, v = k + kFusedChunks * kBN * D * 2,
-                       p = v + kFusedChunks * kBN * D * 2, g = p + kBM * kBN * 2, total = g + kBM * kBN * 2 + 1024;
+                       p = v + kFusedChunks * kBN * D * 2, g = p + kBM * kBN * 2, stage = g + kBM * kBN * 2,
+                       total = stage + kBM * D * 2 + 1024;      // stage: bf16 dQ rows on their way out
   static constexpr uint32_t cS = 0, cDP = 64, cDQ = 128, cDV = 256, cDK = 384, cols = 512;
 };
 
@@ -613,8 +614,8 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar[2];
   __shared__ uint32_t tbase_s;
-  __shared__ int32_t pid_s[2][kBM];
-  const int tid = threadIdx.x, warp = tid >> 5, row = tid & 127, wg = tid >> 7;
+  __shared__ int32_t pid_s[3][kBM];                        // pair ids of the previous, the current and the next tile
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = tid & 127, wg = tid >> 7;
   const int j = blockIdx.x, pq = blockIdx.y;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
@@ -689,30 +690,47 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
     int buf = 0;
     // The dQ rows of a tile are written while the first products of the NEXT tile run on the tensor cores
     // (the accumulator columns are only overwritten by that tile's second batch of MMAs).
-    int prev_pid = 0, prev_nq = 0, prev_nch = -1;              // prev_nch < 0: nothing pending
+    int prev_pid = 0, prev_nq = 0, prev_nch = -1, prev_buf = 0;  // prev_nch < 0: nothing pending
     auto store_dq = [&]() {
-      if (prev_nch < 0) return;
-      // bf16 dQ row per (query, slot); each warpgroup converts and stores half of it.  Later sweeps add to it.
-      bf16* dst = dq_part + ((size_t)pq * dm.N * dm.m + prev_pid) * D + wg * (D / 2);
+      if (prev_nch < 0) return;                                         // uniform over the CTA
       const uint32_t tq = tl + SM::cDQ + wg * (D / 2);
+      bf16* base = dq_part + (size_t)pq * dm.N * dm.m * D;
+      // bf16 rows go through a staging tile (thread = row, 16-byte chunks XOR-swizzled) so that they
+      // leave as whole 256-byte rows, 16 lanes per row: a row-per-thread store would touch 32 lines per
+      // instruction.  Later sweeps (clusters with more keys than one sweep holds) add to the stored rows.
+      unsigned char* stg = c.sm + SM::stage;
 #pragma unroll
       for (int d0 = 0; d0 < D / 2; d0 += 32) {
         float v[32];
         if (prev_nch > 0) tc::tmem_ld32(tq + d0, v);
-        if (row < prev_nq && c.ok) {
 #pragma unroll
-          for (int i = 0; i < 32; i += 8) {
-            float x[8];
+        for (int i = 0; i < 32; i += 8) {
+          uint32_t w[4];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) x[e] = prev_nch > 0 ? v[i + e] * dm.sigma : 0.f;
+          for (int e = 0; e < 4; ++e) {
+            __nv_bfloat162 b2 = prev_nch > 0 ? __floats2bfloat162_rn(v[i + 2 * e] * dm.sigma, v[i + 2 * e + 1] * dm.sigma) : __floats2bfloat162_rn(0.f, 0.f);
+            w[e] = *reinterpret_cast<uint32_t*>(&b2);
+          }
+          const int ck = (wg * (D / 2) + d0 + i) >> 3;
+          *reinterpret_cast<uint4*>(stg + row * 256 + ((ck ^ (row & 15)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      }
+      __syncthreads();
+      if (c.ok) {
+#pragma unroll
+        for (int k = 0; k < kBM / 16; ++k) {                            // 8 warps x 8 steps x 2 rows
+          const int r = warp * 16 + 2 * k + (lane >> 4), ck = lane & 15;
+          if (r < prev_nq) {
+            uint4 val = *reinterpret_cast<const uint4*>(stg + r * 256 + ((ck ^ (r & 15)) << 4));
+            uint4* dst = reinterpret_cast<uint4*>(base + (size_t)pid_s[prev_buf][r] * D + ck * 8);
             if (!first_sweep) {
-              const float4 o0 = ld4(dst + d0 + i), o1 = ld4(dst + d0 + i + 4);
-              x[0] += o0.x; x[1] += o0.y; x[2] += o0.z; x[3] += o0.w; x[4] += o1.x; x[5] += o1.y; x[6] += o1.z; x[7] += o1.w;
-            }
-            uint32_t w[4];
+              const uint4 old = *dst;
+              __nv_bfloat162* a2 = reinterpret_cast<__nv_bfloat162*>(&val);
+              const __nv_bfloat162* o2 = reinterpret_cast<const __nv_bfloat162*>(&old);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) { __nv_bfloat162 b2 = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]); w[e] = *reinterpret_cast<uint32_t*>(&b2); }
-            *reinterpret_cast<uint4*>(dst + d0 + i) = make_uint4(w[0], w[1], w[2], w[3]);
+              for (int e = 0; e < 4; ++e) a2[e] = __floats2bfloat162_rn(__low2float(a2[e]) + __low2float(o2[e]), __high2float(a2[e]) + __high2float(o2[e]));
+            }
+            *dst = val;
           }
         }
       }
@@ -728,23 +746,24 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       const int nq = min(kBM, cur.g1 - cur.t0);
       const int vis = min(KC, max(0, ok[cur.pl + 1] - kc0));            // keys of this sweep that the plane sees
       const int nch = (vis + kBN - 1) / kBN;
+      const int nbuf = buf == 2 ? 0 : buf + 1;
       tile_sts<D, kBM, kFusedThreads>(qreg, c.sm + SM::q, tid);
       tile_sts<D, kBM, kFusedThreads>(oreg, c.sm + SM::dO, tid);
-      if (tid < kBM) pid_s[buf ^ 1][tid] = pidreg;                      // pair ids of the next tile
+      if (tid < kBM) pid_s[nbuf][tid] = pidreg;                         // pair ids of the next tile
       const float L2 = Lreg, dl = dreg;
       const int my_pid = pid_s[buf][row];
       tc::fence_async_smem();
       tc::fence_before_sync();
-      __syncthreads();                                                  // tiles and pid_s[buf ^ 1] visible
+      __syncthreads();                                                  // tiles and pid_s[nbuf] visible
       ZCLK(0)
       bool prefetched = false;
       auto prefetch = [&]() {                                           // gathers of the next tile, pair ids of the one after
         if (prefetched) return;
-        if (nxt.pl < dm.SB) load_rows(nxt, pid_s[buf ^ 1]);
+        if (nxt.pl < dm.SB) load_rows(nxt, pid_s[nbuf]);
         load_pids(nn);
         prefetched = true;
       };
-      for (int ch = 0; ch < nch && c.ok; ++ch) {
+      auto issue_first = [&](int ch) {                                  // S = Q K^T and dP = dO V^T for key chunk ch
         const uint32_t kac = ka + ch * kBN * D * 2, vac = va + ch * kBN * D * 2;
         if (tid == 0) {
           tc::fence_after_sync();
@@ -756,7 +775,12 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
           tc::mma_commit(&c.bar[0]);
         }
         __syncwarp();
-        if (ch == 0) store_dq();                                        // previous tile's rows leave meanwhile
+      };
+      if (nch > 0) issue_first(0);
+      store_dq();                                                       // previous tile's rows leave meanwhile
+      for (int ch = 0; ch < nch && c.ok; ++ch) {
+        const uint32_t kac = ka + ch * kBN * D * 2;
+        if (ch > 0) issue_first(ch);
         ZCLK(1)
         if (!tc::mbar_wait(&c.bar[0], c.ph0)) { c.ok = false; break; }
         c.ph0 ^= 1;
@@ -806,11 +830,10 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
         tc::fence_after_sync();
         ZCLK(5)
       }
-      if (nch == 0) store_dq();                                         // (no product was issued above)
       prefetch();
-      prev_pid = my_pid; prev_nq = nq; prev_nch = nch;
+      prev_pid = my_pid; prev_nq = nq; prev_nch = nch; prev_buf = buf;
       tc::fence_before_sync();
-      cur = nxt; nxt = nn; nn = next_of(nn); buf ^= 1;
+      cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf;
       ZCLK(6)
 #ifdef MUSE_PHASE_CLOCKS
       c.pc[7] += 1;
