@@ -8,6 +8,8 @@
 #include "common.cuh"
 #include "tc05.cuh"
 
+#include <cstdlib>
+
 namespace muse {
 
 typedef __nv_bfloat16 bf16;
@@ -209,7 +211,7 @@ template <int D>
 __global__ void __launch_bounds__(128)
 k_ret_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, const bf16* __restrict__ Vp,
              const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
-             bf16* __restrict__ o_part, float* __restrict__ l_part, int* __restrict__ status) {
+             bf16* __restrict__ o_part, float* __restrict__ l_part, int min_cluster_keys, int* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar[2];
   __shared__ uint32_t tbase_s;
@@ -223,6 +225,7 @@ k_ret_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, c
   if (g0 + sub * kTcM >= g1) return;                     // no pair tile for this split (before any TMEM allocation)
   const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const int k0 = ok[0], k1 = ok[pl + 1];
+  if (ok[dm.SB] - k0 < min_cluster_keys) return;         // short clusters are handled by the cluster-resident kernel
   TcCtx c;
   tc_setup<D>(c, sm_raw, bar, &tbase_s, tid);
   const bf16* Qb = Q + (size_t)pq * dm.N * D;
@@ -260,6 +263,254 @@ k_ret_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, c
   tc_teardown<D>(c, tid, status);
 }
 
+// ---- exact retrieval, cluster-resident version (D = 128, clusters with at most 128 visible keys) -------
+// One CTA per (key cluster j, head): the cluster's keys and values stay in shared memory (two chunks
+// of 64) while the CTA walks the retrieving (query, slot) pairs of every plane in tiles of 128.  All
+// logits of a tile come from one batch of MMAs, so the softmax needs no running rescale; the Q rows
+// of the next tile are gathered (registers) and the finished rows of the previous tile are written
+// (staged, whole 256-byte rows) while the tensor core works on the current one.
+constexpr int kRcThreads = 256, kRcKeys = 128;
+
+struct RcSmem {
+  static constexpr int D = 128;
+  static constexpr int q = 0, k = q + kTcM * D * 2, v = k + kRcKeys * D * 2, p = v + kRcKeys * D * 2,
+                       stage = p + 2 * kTcM * kTcN * 2, total = stage + kTcM * D * 2 + 1024;
+  static constexpr uint32_t cS = 0, cO = 128, cols = 256;
+};
+
+__global__ void __launch_bounds__(kRcThreads, 1)
+k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, const bf16* __restrict__ Vp,
+                     const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
+                     bf16* __restrict__ o_part, float* __restrict__ l_part, int* __restrict__ status) {
+  typedef RcSmem SM;
+  constexpr int D = SM::D;
+  extern __shared__ __align__(1024) unsigned char sm_raw[];
+  __shared__ uint64_t bar[2];
+  __shared__ uint32_t tbase_s;
+  __shared__ int32_t pid_s[3][kTcM];                       // pair ids of the previous, the current and the next tile
+  __shared__ float mx_s[2][kTcM], sum_s[2][kTcM];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = tid & 127, wg = tid >> 7;
+  const int j = blockIdx.x, pq = blockIdx.y;
+  const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
+  const int nkeys = dm.SB * dm.Ck;
+  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + j;                // group of plane pl: go[pl * Ck], go[pl * Ck + 1]
+  const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
+  const int k0 = ok[0], kall = ok[dm.SB];
+  if (kall - k0 > kRcKeys) return;                          // long clusters take the streaming kernel
+  bool any_pair = false;
+  for (int pl = 0; pl < dm.SB; ++pl) any_pair |= go[(size_t)pl * dm.Ck + 1] > go[(size_t)pl * dm.Ck];
+  if (!any_pair) return;
+
+  unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
+  if (warp == 0) tc::tmem_alloc(&tbase_s, SM::cols);
+  if (tid == 0) { tc::mbar_init(&bar[0], 1); tc::mbar_init(&bar[1], 1); tc::mbar_init_fence(); }
+  const bf16* Qb = Q + (size_t)pq * dm.N * D;
+  const bf16* Kb = Kp + (size_t)pk * dm.N * D;
+  const bf16* Vb = Vp + (size_t)pk * dm.N * D;
+  const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
+  // the cluster's keys (K-major for S = Q K^T) and values (MN-major for O = P V), two chunks of 64
+  for (int ch = 0; ch < 2; ++ch) {
+    const int n = min(kTcN, max(0, kall - k0 - ch * kTcN));
+    for (int e = tid; e < kTcN * (D / 8); e += kRcThreads) {
+      const int r = e / (D / 8), ck = e % (D / 8);
+      uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+      if (r < n) {
+        a = reinterpret_cast<const uint4*>(Kb + (size_t)(k0 + ch * kTcN + r) * D)[ck];
+        b = reinterpret_cast<const uint4*>(Vb + (size_t)(k0 + ch * kTcN + r) * D)[ck];
+      }
+      const uint32_t off = ch * kTcN * D * 2 + (ck >> 3) * kTcN * 128 + tc::sw128_off(r, ck & 7);
+      *reinterpret_cast<uint4*>(sm + SM::k + off) = a;
+      *reinterpret_cast<uint4*>(sm + SM::v + off) = b;
+    }
+  }
+  tc::fence_async_smem();
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tbase = tbase_s, tl = tbase + ((uint32_t)((warp & 3) * 32) << 16);
+  const uint32_t qa = tc::smem_u32(sm + SM::q), ka = tc::smem_u32(sm + SM::k), va = tc::smem_u32(sm + SM::v), pa = tc::smem_u32(sm + SM::p);
+  const float scale2 = dm.sigma * 1.4426950408889634f;
+  uint32_t ph0 = 0, ph1 = 0;
+  bool ok_ = true;
+
+  struct Item { int pl, t0, g1; };
+  auto first_from = [&](int pl) {
+    Item it; it.pl = pl; it.t0 = 0; it.g1 = 0;
+    while (it.pl < dm.SB && go[(size_t)it.pl * dm.Ck + 1] <= go[(size_t)it.pl * dm.Ck]) ++it.pl;
+    if (it.pl < dm.SB) { it.t0 = go[(size_t)it.pl * dm.Ck]; it.g1 = go[(size_t)it.pl * dm.Ck + 1]; }
+    return it;
+  };
+  auto next_of = [&](const Item& a) {
+    if (a.pl >= dm.SB) return a;
+    if (a.t0 + kTcM < a.g1) { Item it = a; it.t0 += kTcM; return it; }
+    return first_from(a.pl + 1);
+  };
+  uint4 qreg[kTcM * (D / 8) / kRcThreads];                 // the next tile's Q rows between their loads and their stores
+  int pidreg = 0;
+  auto load_pids = [&](const Item& it) {
+    if (tid < kTcM) pidreg = (it.pl < dm.SB && it.t0 + tid < it.g1) ? __ldg(pr + it.t0 + tid) : 0;
+  };
+  auto load_rows = [&](const Item& it, const int32_t* pid) {
+    const int nq = min(kTcM, it.g1 - it.t0);
+#pragma unroll
+    for (int k = 0; k < kTcM * (D / 8) / kRcThreads; ++k) {
+      const int e = tid + kRcThreads * k, r = e / (D / 8), ck = e % (D / 8);
+      qreg[k] = r < nq ? __ldg(reinterpret_cast<const uint4*>(Qb + (size_t)(pid[r] / dm.m) * D) + ck) : make_uint4(0u, 0u, 0u, 0u);
+    }
+  };
+  // finished rows of the previous tile: normalised, bf16, staged, then stored 16 lanes per row
+  int prev_nq = 0, prev_buf = 0;
+  float prev_inv = 0.f, prev_lse = 0.f;
+  bool pending = false;
+  auto store_prev = [&]() {
+    if (!pending) return;                                 // uniform over the CTA
+    unsigned char* stg = sm + SM::stage;
+#pragma unroll
+    for (int d0 = 0; d0 < D / 2; d0 += 32) {
+      float v[32];
+      tc::tmem_ld32(tl + SM::cO + wg * (D / 2) + d0, v);
+#pragma unroll
+      for (int i = 0; i < 32; i += 8) {
+        uint32_t w[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          __nv_bfloat162 b2 = __floats2bfloat162_rn(v[i + 2 * e] * prev_inv, v[i + 2 * e + 1] * prev_inv);
+          w[e] = *reinterpret_cast<uint32_t*>(&b2);
+        }
+        const int ck = (wg * (D / 2) + d0 + i) >> 3;
+        *reinterpret_cast<uint4*>(stg + row * 256 + ((ck ^ (row & 15)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+    }
+    if (wg == 0 && row < prev_nq && ok_) l_part[(size_t)pq * dm.N * dm.m + pid_s[prev_buf][row]] = prev_lse;
+    __syncthreads();
+    if (ok_) {
+      bf16* base = o_part + (size_t)pq * dm.N * dm.m * D;
+#pragma unroll
+      for (int k = 0; k < kTcM / 16; ++k) {
+        const int r = warp * 16 + 2 * k + (lane >> 4), ck = lane & 15;
+        if (r < prev_nq)
+          *reinterpret_cast<uint4*>(base + (size_t)pid_s[prev_buf][r] * D + ck * 8) =
+              *reinterpret_cast<const uint4*>(stg + r * 256 + ((ck ^ (r & 15)) << 4));
+      }
+    }
+    pending = false;
+  };
+
+  Item cur = first_from(0), nxt = next_of(cur), nn = next_of(nxt);
+  load_pids(cur);
+  if (tid < kTcM) pid_s[0][tid] = pidreg;
+  load_pids(nxt);
+  __syncthreads();
+  if (cur.pl < dm.SB) load_rows(cur, pid_s[0]);
+  int buf = 0;
+  while (cur.pl < dm.SB && ok_) {
+    const int nq = min(kTcM, cur.g1 - cur.t0);
+    const int vis = ok[cur.pl + 1] - k0;                    // keys the plane sees (<= 128)
+    const int nch = (vis + kTcN - 1) / kTcN;
+    const int nbuf = buf == 2 ? 0 : buf + 1;
+#pragma unroll
+    for (int k = 0; k < kTcM * (D / 8) / kRcThreads; ++k) {
+      const int e = tid + kRcThreads * k, r = e / (D / 8), ck = e % (D / 8);
+      *reinterpret_cast<uint4*>(sm + SM::q + (ck >> 3) * kTcM * 128 + tc::sw128_off(r, ck & 7)) = qreg[k];
+    }
+    if (tid < kTcM) pid_s[nbuf][tid] = pidreg;              // pair ids of the next tile
+    tc::fence_async_smem();
+    tc::fence_before_sync();
+    __syncthreads();
+    if (tid == 0 && nch > 0) {
+      tc::fence_after_sync();
+      const uint32_t idesc = tc::idesc_bf16(kTcM, kTcN, 0, 0);
+      for (int ch = 0; ch < nch; ++ch) {
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks)
+          tc::mma_bf16_ss(tbase + SM::cS + ch * kTcN, tc::smem_desc_sw128(qa + (ks / 4) * kTcM * 128 + (ks % 4) * 32, 16, 1024),
+                          tc::smem_desc_sw128(ka + ch * kTcN * D * 2 + (ks / 4) * kTcN * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
+      }
+      tc::mma_commit(&bar[0]);
+    }
+    __syncwarp();
+    if (nxt.pl < dm.SB) load_rows(nxt, pid_s[nbuf]);        // gathers fly while this tile is processed
+    load_pids(nn);
+    store_prev();                                           // the previous tile's rows leave meanwhile
+    float M = -INFINITY, l = 0.f;
+    if (nch > 0) {
+      if (!tc::mbar_wait(&bar[0], ph0)) ok_ = false;
+      ph0 ^= 1;
+      tc::fence_after_sync();
+      // softmax over up to 128 keys: warpgroup = key chunk; the two halves of a row meet through shared memory
+      float sv[kTcN];
+      const int visc = vis - wg * kTcN;                     // visible columns of this warpgroup's chunk
+      float mx = -INFINITY;
+      if (wg < nch) {
+        tc::tmem_ld32(tl + SM::cS + wg * kTcN, *reinterpret_cast<float(*)[32]>(&sv[0]));
+        tc::tmem_ld32(tl + SM::cS + wg * kTcN + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+#pragma unroll
+        for (int i = 0; i < kTcN; ++i) { sv[i] = i < visc ? sv[i] * scale2 : -INFINITY; mx = fmaxf(mx, sv[i]); }
+      }
+      mx_s[wg][row] = mx;
+      __syncthreads();
+      M = fmaxf(mx_s[0][row], mx_s[1][row]);
+      float rs = 0.f;
+      if (wg < nch) {
+        const float base = M == -INFINITY ? 0.f : M;
+        uint32_t pk[kTcN / 2];
+#pragma unroll
+        for (int i = 0; i < kTcN; i += 2) {
+          __nv_bfloat162 b = __floats2bfloat162_rn(tc::fast_exp2(sv[i] - base), tc::fast_exp2(sv[i + 1] - base));
+          rs += __low2float(b) + __high2float(b);            // the rounded values, as the P V product sees them
+          pk[i / 2] = *reinterpret_cast<uint32_t*>(&b);
+        }
+#pragma unroll
+        for (int ch8 = 0; ch8 < kTcN / 8; ++ch8)
+          *reinterpret_cast<uint4*>(sm + SM::p + wg * kTcM * kTcN * 2 + tc::sw128_off(row, ch8)) =
+              make_uint4(pk[ch8 * 4], pk[ch8 * 4 + 1], pk[ch8 * 4 + 2], pk[ch8 * 4 + 3]);
+      }
+      sum_s[wg][row] = rs;
+      tc::fence_async_smem();
+      tc::fence_before_sync();
+      __syncthreads();
+      if (tid == 0) {
+        tc::fence_after_sync();
+        const uint32_t idesc = tc::idesc_bf16(kTcM, D, 0, 1);
+        for (int ch = 0; ch < nch; ++ch) {
+#pragma unroll
+          for (int ks = 0; ks < kTcN / 16; ++ks)
+            tc::mma_bf16_ss(tbase + SM::cO, tc::smem_desc_sw128(pa + ch * kTcM * kTcN * 2 + ks * 32, 16, 1024),
+                            tc::smem_desc_sw128(va + ch * kTcN * D * 2 + ks * 16 * 128, kTcN * 128, 1024), idesc, ch > 0 || ks > 0);
+        }
+        tc::mma_commit(&bar[1]);
+      }
+      __syncwarp();
+      l = sum_s[0][row] + sum_s[1][row];
+      if (!tc::mbar_wait(&bar[1], ph1)) ok_ = false;
+      ph1 ^= 1;
+      tc::fence_after_sync();
+    }
+    // what the deferred store needs: 1 / l and the log-sum-exp of the row (natural log)
+    prev_inv = l > 0.f ? 1.f / l : 0.f;
+    prev_lse = l > 0.f ? (M + log2f(l)) * 0.6931471805599453f : -INFINITY;
+    prev_nq = nq; prev_buf = buf; pending = true;
+    if (nch == 0) {
+      // nothing visible (possible with forced selections): rows of zeros, done here because the accumulator holds no data
+      if (row < nq && ok_) {
+        const size_t pid = (size_t)pq * dm.N * dm.m + pid_s[buf][row];
+        uint4* dst = reinterpret_cast<uint4*>(o_part + pid * D + wg * (D / 2));
+#pragma unroll
+        for (int i = 0; i < D / 16; ++i) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (wg == 0) l_part[pid] = -INFINITY;
+      }
+      pending = false;
+    }
+    tc::fence_before_sync();
+    cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf;
+  }
+  store_prev();
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tbase, SM::cols);
+  if (!ok_ && tid == 0) atomicExch(status, 1);
+}
+
 int local_fwd_tc(const Dims& d, const void* Q, const void* K, const void* V, float* o_loc, float* lse_loc, int* status,
                  cudaStream_t st) {
   const int pq = d.B * d.Hq;
@@ -279,13 +530,23 @@ int local_fwd_tc(const Dims& d, const void* Q, const void* K, const void* V, flo
 int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
                const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st) {
   dim3 grid(d.Ck, d.SB * kRetFwdSplit, d.B * d.Hq);
+  int min_keys = 0;                      // the streaming kernel takes every cluster ...
+  if (d.D == 128 && getenv("MUSE_RET_FWD_STREAM") == nullptr) {
+    // ... except, at D = 128, those whose keys fit the cluster-resident kernel
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_cluster_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, RcSmem::total));
+    prof_mark("k_ret_fwd_cluster_tc", st);
+    k_ret_fwd_cluster_tc<<<dim3(d.Ck, d.B * d.Hq), kRcThreads, RcSmem::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k,
+                                                                                 goff, pairs, (bf16*)o_part, l_part, status);
+    MUSE_LAUNCH_OK();
+    min_keys = kRcKeys + 1;
+  }
   prof_mark("k_ret_fwd_tc", st);
   if (d.D == 128) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdTcSmem<128>::total));
-    k_ret_fwd_tc<128><<<grid, 128, FwdTcSmem<128>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs, (bf16*)o_part, l_part, status);
+    k_ret_fwd_tc<128><<<grid, 128, FwdTcSmem<128>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs, (bf16*)o_part, l_part, min_keys, status);
   } else {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdTcSmem<64>::total));
-    k_ret_fwd_tc<64><<<grid, 128, FwdTcSmem<64>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs, (bf16*)o_part, l_part, status);
+    k_ret_fwd_tc<64><<<grid, 128, FwdTcSmem<64>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs, (bf16*)o_part, l_part, min_keys, status);
   }
   MUSE_LAUNCH_OK();
   return MUSE_OK;
