@@ -263,12 +263,14 @@ k_ret_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, c
   tc_teardown<D>(c, tid, status);
 }
 
-// ---- exact retrieval, cluster-resident version (D = 128, clusters with at most 128 visible keys) -------
-// One CTA per (key cluster j, head): the cluster's keys and values stay in shared memory (two chunks
-// of 64) while the CTA walks the retrieving (query, slot) pairs of every plane in tiles of 128.  All
-// logits of a tile come from one batch of MMAs, so the softmax needs no running rescale; the Q rows
+// ---- exact retrieval, cluster-resident version (D = 128) ---------------------------------------------
+// One CTA per (key cluster j, head): 128 of the cluster's keys and values stay in shared memory (two
+// chunks of 64) while the CTA walks the retrieving (query, slot) pairs of every plane in tiles of 128.
+// All logits of a tile come from one batch of MMAs, so the softmax needs no running rescale; the Q rows
 // of the next tile are gathered (registers) and the finished rows of the previous tile are written
-// (staged, whole 256-byte rows) while the tensor core works on the current one.
+// (staged, whole 256-byte rows) while the tensor core works on the current one.  A cluster with more
+// than 128 visible keys takes further sweeps, whose partial results are merged into the stored rows by
+// their log-sum-exp weights.
 constexpr int kRcThreads = 256, kRcKeys = 128;
 
 struct RcSmem {
@@ -288,7 +290,7 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   __shared__ uint64_t bar[2];
   __shared__ uint32_t tbase_s;
   __shared__ int32_t pid_s[3][kTcM];                       // pair ids of the previous, the current and the next tile
-  __shared__ float mx_s[2][kTcM], sum_s[2][kTcM];
+  __shared__ float mx_s[2][kTcM], sum_s[2][kTcM], wold_s[kTcM], wnew_s[kTcM];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = tid & 127, wg = tid >> 7;
   const int j = blockIdx.x, pq = blockIdx.y;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
@@ -296,7 +298,6 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   const int32_t* go = goff + (size_t)pq * (nkeys + 1) + j;                // group of plane pl: go[pl * Ck], go[pl * Ck + 1]
   const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const int k0 = ok[0], kall = ok[dm.SB];
-  if (kall - k0 > kRcKeys) return;                          // long clusters take the streaming kernel
   bool any_pair = false;
   for (int pl = 0; pl < dm.SB; ++pl) any_pair |= go[(size_t)pl * dm.Ck + 1] > go[(size_t)pl * dm.Ck];
   if (!any_pair) return;
@@ -308,21 +309,6 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   const bf16* Kb = Kp + (size_t)pk * dm.N * D;
   const bf16* Vb = Vp + (size_t)pk * dm.N * D;
   const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
-  // the cluster's keys (K-major for S = Q K^T) and values (MN-major for O = P V), two chunks of 64
-  for (int ch = 0; ch < 2; ++ch) {
-    const int n = min(kTcN, max(0, kall - k0 - ch * kTcN));
-    for (int e = tid; e < kTcN * (D / 8); e += kRcThreads) {
-      const int r = e / (D / 8), ck = e % (D / 8);
-      uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
-      if (r < n) {
-        a = reinterpret_cast<const uint4*>(Kb + (size_t)(k0 + ch * kTcN + r) * D)[ck];
-        b = reinterpret_cast<const uint4*>(Vb + (size_t)(k0 + ch * kTcN + r) * D)[ck];
-      }
-      const uint32_t off = ch * kTcN * D * 2 + (ck >> 3) * kTcN * 128 + tc::sw128_off(r, ck & 7);
-      *reinterpret_cast<uint4*>(sm + SM::k + off) = a;
-      *reinterpret_cast<uint4*>(sm + SM::v + off) = b;
-    }
-  }
   tc::fence_async_smem();
   tc::fence_before_sync();
   __syncthreads();
@@ -334,9 +320,11 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   bool ok_ = true;
 
   struct Item { int pl, t0, g1; };
+  int kc0 = k0;                                             // first key of the current sweep
+  bool first_sweep = true;
   auto first_from = [&](int pl) {
     Item it; it.pl = pl; it.t0 = 0; it.g1 = 0;
-    while (it.pl < dm.SB && go[(size_t)it.pl * dm.Ck + 1] <= go[(size_t)it.pl * dm.Ck]) ++it.pl;
+    while (it.pl < dm.SB && (go[(size_t)it.pl * dm.Ck + 1] <= go[(size_t)it.pl * dm.Ck] || (!first_sweep && ok[it.pl + 1] <= kc0))) ++it.pl;
     if (it.pl < dm.SB) { it.t0 = go[(size_t)it.pl * dm.Ck]; it.g1 = go[(size_t)it.pl * dm.Ck + 1]; }
     return it;
   };
@@ -361,7 +349,7 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   // finished rows of the previous tile: normalised, bf16, staged, then stored 16 lanes per row
   int prev_nq = 0, prev_buf = 0;
   float prev_inv = 0.f, prev_lse = 0.f;
-  bool pending = false;
+  bool pending = false, prev_first = true;
   auto store_prev = [&]() {
     if (!pending) return;                                 // uniform over the CTA
     unsigned char* stg = sm + SM::stage;
@@ -381,21 +369,63 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
         *reinterpret_cast<uint4*>(stg + row * 256 + ((ck ^ (row & 15)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
       }
     }
-    if (wg == 0 && row < prev_nq && ok_) l_part[(size_t)pq * dm.N * dm.m + pid_s[prev_buf][row]] = prev_lse;
+    if (wg == 0 && row < prev_nq && ok_) {
+      float* lp = l_part + (size_t)pq * dm.N * dm.m + pid_s[prev_buf][row];
+      if (prev_first) {
+        *lp = prev_lse;
+      } else {
+        // merge with what earlier sweeps stored: weights exp(L_old - L), exp(L_new - L), L = log(e^L_old + e^L_new)
+        const float lo = *lp, ln = prev_lse, mxl = fmaxf(lo, ln);
+        const float eo = lo == -INFINITY ? 0.f : __expf(lo - mxl), en = ln == -INFINITY ? 0.f : __expf(ln - mxl);
+        const float tot = eo + en;
+        wold_s[row] = tot > 0.f ? eo / tot : 0.f;
+        wnew_s[row] = tot > 0.f ? en / tot : 0.f;
+        *lp = tot > 0.f ? mxl + __logf(tot) : -INFINITY;
+      }
+    }
     __syncthreads();
     if (ok_) {
       bf16* base = o_part + (size_t)pq * dm.N * dm.m * D;
 #pragma unroll
       for (int k = 0; k < kTcM / 16; ++k) {
         const int r = warp * 16 + 2 * k + (lane >> 4), ck = lane & 15;
-        if (r < prev_nq)
-          *reinterpret_cast<uint4*>(base + (size_t)pid_s[prev_buf][r] * D + ck * 8) =
-              *reinterpret_cast<const uint4*>(stg + r * 256 + ((ck ^ (r & 15)) << 4));
+        if (r < prev_nq) {
+          uint4 val = *reinterpret_cast<const uint4*>(stg + r * 256 + ((ck ^ (r & 15)) << 4));
+          uint4* dst = reinterpret_cast<uint4*>(base + (size_t)pid_s[prev_buf][r] * D + ck * 8);
+          if (!prev_first) {
+            const uint4 old = *dst;
+            const float wo = wold_s[r], wn = wnew_s[r];
+            __nv_bfloat162* a2 = reinterpret_cast<__nv_bfloat162*>(&val);
+            const __nv_bfloat162* o2 = reinterpret_cast<const __nv_bfloat162*>(&old);
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              a2[e] = __floats2bfloat162_rn(wn * __low2float(a2[e]) + wo * __low2float(o2[e]), wn * __high2float(a2[e]) + wo * __high2float(o2[e]));
+          }
+          *dst = val;
+        }
       }
     }
     pending = false;
   };
 
+  for (; (kc0 < kall || first_sweep) && ok_; kc0 += kRcKeys, first_sweep = false) {
+  __syncthreads();                                          // the previous sweep is done with the key / value tiles
+  // the cluster's keys (K-major for S = Q K^T) and values (MN-major for O = P V), two chunks of 64
+  for (int ch = 0; ch < 2; ++ch) {
+    const int n = min(kTcN, max(0, kall - kc0 - ch * kTcN));
+    for (int e = tid; e < kTcN * (D / 8); e += kRcThreads) {
+      const int r = e / (D / 8), ck = e % (D / 8);
+      uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+      if (r < n) {
+        a = reinterpret_cast<const uint4*>(Kb + (size_t)(kc0 + ch * kTcN + r) * D)[ck];
+        b = reinterpret_cast<const uint4*>(Vb + (size_t)(kc0 + ch * kTcN + r) * D)[ck];
+      }
+      const uint32_t off = ch * kTcN * D * 2 + (ck >> 3) * kTcN * 128 + tc::sw128_off(r, ck & 7);
+      *reinterpret_cast<uint4*>(sm + SM::k + off) = a;
+      *reinterpret_cast<uint4*>(sm + SM::v + off) = b;
+    }
+  }
+  tc::fence_async_smem();
   Item cur = first_from(0), nxt = next_of(cur), nn = next_of(nxt);
   load_pids(cur);
   if (tid < kTcM) pid_s[0][tid] = pidreg;
@@ -405,7 +435,7 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   int buf = 0;
   while (cur.pl < dm.SB && ok_) {
     const int nq = min(kTcM, cur.g1 - cur.t0);
-    const int vis = ok[cur.pl + 1] - k0;                    // keys the plane sees (<= 128)
+    const int vis = min(kRcKeys, max(0, ok[cur.pl + 1] - kc0));   // keys of this sweep that the plane sees
     const int nch = (vis + kTcN - 1) / kTcN;
     const int nbuf = buf == 2 ? 0 : buf + 1;
 #pragma unroll
@@ -489,7 +519,7 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
     // what the deferred store needs: 1 / l and the log-sum-exp of the row (natural log)
     prev_inv = l > 0.f ? 1.f / l : 0.f;
     prev_lse = l > 0.f ? (M + log2f(l)) * 0.6931471805599453f : -INFINITY;
-    prev_nq = nq; prev_buf = buf; pending = true;
+    prev_nq = nq; prev_buf = buf; pending = true; prev_first = first_sweep;
     if (nch == 0) {
       // nothing visible (possible with forced selections): rows of zeros, done here because the accumulator holds no data
       if (row < nq && ok_) {
@@ -505,6 +535,7 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
     cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf;
   }
   store_prev();
+  }
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tbase, SM::cols);
@@ -530,15 +561,14 @@ int local_fwd_tc(const Dims& d, const void* Q, const void* K, const void* V, flo
 int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
                const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st) {
   dim3 grid(d.Ck, d.SB * kRetFwdSplit, d.B * d.Hq);
-  int min_keys = 0;                      // the streaming kernel takes every cluster ...
+  const int min_keys = 0;
   if (d.D == 128 && getenv("MUSE_RET_FWD_STREAM") == nullptr) {
-    // ... except, at D = 128, those whose keys fit the cluster-resident kernel
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_cluster_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, RcSmem::total));
     prof_mark("k_ret_fwd_cluster_tc", st);
     k_ret_fwd_cluster_tc<<<dim3(d.Ck, d.B * d.Hq), kRcThreads, RcSmem::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k,
                                                                                  goff, pairs, (bf16*)o_part, l_part, status);
     MUSE_LAUNCH_OK();
-    min_keys = kRcKeys + 1;
+    return MUSE_OK;
   }
   prof_mark("k_ret_fwd_tc", st);
   if (d.D == 128) {
