@@ -2,8 +2,9 @@
 // products from tcgen05 MMAs.  The centres are fp32; they enter the MMA as a bf16 hi + lo pair
 // (two accumulating products), which keeps ~16 mantissa bits so that the discrete assignment
 // agrees with an fp64 evaluation except at genuine near-ties (Appendix "Balanced Assignment":
-// the |x|^2 term cancels between centres).  One CTA = 128 points, one thread per point scans
-// the distance row chunk by chunk straight out of tensor memory.
+// the |x|^2 term cancels between centres).  One CTA = 128 points; the distance rows are scanned
+// straight out of tensor memory while the next centre tile is being multiplied.
+#include <cuda.h>
 #include "common.cuh"
 #include "tc05.cuh"
 
@@ -22,91 +23,122 @@ __global__ void k_split_centres(const float* __restrict__ c, long long n, bf16* 
   lo[e] = __float2bfloat16_rn(x - __bfloat162float(h));
 }
 
+// Warp roles: warps 0-7 read the distance rows out of tensor memory (two warpgroups, 64 columns each),
+// warp 8 feeds the centre tiles by TMA through a ring, warp 9 issues the MMAs into two alternating
+// accumulator buffers, so that the arg-min sweep of one centre tile overlaps the products of the next.
+constexpr int kAtThreads = 320, kAtEpi = 256;
+
+struct AtBars { uint64_t full[4], empty[4], tfull[2], tempty[2], xbar; };
+
 template <int D>
-__global__ void __launch_bounds__(128)
-k_assign_tc(const bf16* __restrict__ X, int N, int C, const bf16* __restrict__ chi, const bf16* __restrict__ clo,
-            const float* __restrict__ cnorm, int32_t* __restrict__ assign, int* __restrict__ status) {
+__global__ void __launch_bounds__(kAtThreads, 1)
+k_assign_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_hi, const __grid_constant__ CUtensorMap tm_lo,
+            int N, int C, int ns, const float* __restrict__ cnorm, int32_t* __restrict__ assign, int* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char sm_raw[];
-  __shared__ uint64_t bar;
+  __shared__ AtBars bars;
   __shared__ uint32_t tbase_s;
-  __shared__ float cn[kAtCols];
-  constexpr int kX = kAtRows * D * 2, kC = kAtCols * D * 2;
+  __shared__ float best_s[kAtRows];
+  __shared__ int idx_s[kAtRows];
+  constexpr int kX = kAtRows * D * 2, kC = kAtCols * D * 2, kStage = 2 * kC;     // stage = hi tile | lo tile
   unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
-  unsigned char *Xs = sm, *Hs = sm + kX, *Ls = Hs + kC;
+  unsigned char* Xs = sm;
+  unsigned char* ring = sm + kX;
+  float* cn = reinterpret_cast<float*>(ring + ns * kStage);                      // |c|^2 of every centre of this problem
   const int tid = threadIdx.x, warp = tid >> 5, prob = blockIdx.y, row0 = blockIdx.x * kAtRows;
-  if (warp == 0) tc::tmem_alloc(&tbase_s, kAtCols);
-  if (tid == 0) { tc::mbar_init(&bar, 1); tc::mbar_init_fence(); }
-  const bf16* Xp = X + (size_t)prob * N * D;
-  const bf16* hp = chi + (size_t)prob * C * D;
-  const bf16* lp = clo + (size_t)prob * C * D;
-  const float* cnp = cnorm + (size_t)prob * C;
-  constexpr int CPR = D / 8;
-  for (int e = tid; e < kAtRows * CPR; e += 128) {
-    const int r = e / CPR, ck = e % CPR;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (row0 + r < N) v = reinterpret_cast<const uint4*>(Xp + (size_t)(row0 + r) * D)[ck];
-    *reinterpret_cast<uint4*>(Xs + (ck >> 3) * kAtRows * 128 + tc::sw128_off(r, ck & 7)) = v;
+  const int NT = (C + kAtCols - 1) / kAtCols;
+  if (warp == 0) tc::tmem_alloc(&tbase_s, 2 * kAtCols);
+  if (tid == 0) {
+    for (int s = 0; s < 4; ++s) { tc::mbar_init(&bars.full[s], 1); tc::mbar_init(&bars.empty[s], 1); }
+    for (int b = 0; b < 2; ++b) { tc::mbar_init(&bars.tfull[b], 1); tc::mbar_init(&bars.tempty[b], kAtEpi); }
+    tc::mbar_init(&bars.xbar, 1);
+    tc::mbar_init_fence();
   }
+  for (int c = tid; c < NT * kAtCols; c += kAtThreads) cn[c] = c < C ? cnorm[(size_t)prob * C + c] : INFINITY;
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
-  const uint32_t tbase = tbase_s, tlane = tbase + ((uint32_t)(warp * 32) << 16);
-  uint32_t ph = 0;
+  const uint32_t tbase = tbase_s;
   bool ok = true;
-  float best = INFINITY;
-  int bidx = 0x7fffffff;
-  for (int c0 = 0; c0 < C && ok; c0 += kAtCols) {
-    for (int e = tid; e < kAtCols * CPR; e += 128) {
-      const int r = e / CPR, ck = e % CPR;
-      uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
-      if (c0 + r < C) {
-        a = reinterpret_cast<const uint4*>(hp + (size_t)(c0 + r) * D)[ck];
-        b = reinterpret_cast<const uint4*>(lp + (size_t)(c0 + r) * D)[ck];
+
+  if (warp == 8) {
+    if (tid == 8 * 32) {                                   // ---- producer
+      tc::mbar_expect_tx(&bars.xbar, kX);
+      for (int g = 0; g < D / 64; ++g) tc::tma_load_2d(Xs + g * kAtRows * 128, &tm_x, 64 * g, prob * N + row0, &bars.xbar);
+      for (int t = 0; t < NT && ok; ++t) {
+        const int s = t % ns;
+        if (!tc::mbar_wait(&bars.empty[s], ((t / ns) & 1) ^ 1)) { ok = false; break; }
+        tc::mbar_expect_tx(&bars.full[s], kStage);
+        unsigned char* st = ring + s * kStage;
+        for (int g = 0; g < D / 64; ++g) {
+          tc::tma_load_2d(st + g * kAtCols * 128, &tm_hi, 64 * g, prob * C + t * kAtCols, &bars.full[s]);
+          tc::tma_load_2d(st + kC + g * kAtCols * 128, &tm_lo, 64 * g, prob * C + t * kAtCols, &bars.full[s]);
+        }
       }
-      const uint32_t off = (ck >> 3) * kAtCols * 128 + tc::sw128_off(r, ck & 7);
-      *reinterpret_cast<uint4*>(Hs + off) = a;
-      *reinterpret_cast<uint4*>(Ls + off) = b;
     }
-    cn[tid] = c0 + tid < C ? cnp[c0 + tid] : INFINITY;
-    tc::fence_async_smem();
-    tc::fence_before_sync();
-    __syncthreads();
-    if (tid == 0) {
-      tc::fence_after_sync();
+  } else if (warp == 9) {
+    if (tid == 9 * 32) {                                   // ---- MMA issuer
       const uint32_t idesc = tc::idesc_bf16(kAtRows, kAtCols, 0, 0);
-      const uint32_t xa = tc::smem_u32(Xs), ha = tc::smem_u32(Hs), la = tc::smem_u32(Ls);
+      const uint32_t xa = tc::smem_u32(Xs);
+      if (!tc::mbar_wait(&bars.xbar, 0)) ok = false;
+      for (int t = 0; t < NT && ok; ++t) {
+        const int s = t % ns, b = t & 1;
+        if (!tc::mbar_wait(&bars.tempty[b], ((t >> 1) & 1) ^ 1)) { ok = false; break; }
+        if (!tc::mbar_wait(&bars.full[s], (t / ns) & 1)) { ok = false; break; }
+        tc::fence_after_sync();
+        const uint32_t ha = tc::smem_u32(ring + s * kStage), la = ha + kC;
 #pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks)
-        tc::mma_bf16_ss(tbase, tc::smem_desc_sw128(xa + (ks / 4) * kAtRows * 128 + (ks % 4) * 32, 16, 1024),
-                        tc::smem_desc_sw128(ha + (ks / 4) * kAtCols * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
+        for (int ks = 0; ks < D / 16; ++ks)
+          tc::mma_bf16_ss(tbase + b * kAtCols, tc::smem_desc_sw128(xa + (ks / 4) * kAtRows * 128 + (ks % 4) * 32, 16, 1024),
+                          tc::smem_desc_sw128(ha + (ks / 4) * kAtCols * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
 #pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks)
-        tc::mma_bf16_ss(tbase, tc::smem_desc_sw128(xa + (ks / 4) * kAtRows * 128 + (ks % 4) * 32, 16, 1024),
-                        tc::smem_desc_sw128(la + (ks / 4) * kAtCols * 128 + (ks % 4) * 32, 16, 1024), idesc, 1);
-      tc::mma_commit(&bar);
-    }
-    if (!tc::mbar_wait(&bar, ph)) ok = false;
-    ph ^= 1;
-    tc::fence_after_sync();
-#pragma unroll
-    for (int q = 0; q < kAtCols / 32; ++q) {
-      float v[32];
-      tc::tmem_ld32(tlane + 32 * q, v);
-#pragma unroll
-      for (int k = 0; k < 32; ++k) {
-        const float dist = fmaf(-2.f, v[k], cn[32 * q + k]);
-        if (dist < best) { best = dist; bidx = c0 + 32 * q + k; }     // ascending index: ties keep the lower
+        for (int ks = 0; ks < D / 16; ++ks)
+          tc::mma_bf16_ss(tbase + b * kAtCols, tc::smem_desc_sw128(xa + (ks / 4) * kAtRows * 128 + (ks % 4) * 32, 16, 1024),
+                          tc::smem_desc_sw128(la + (ks / 4) * kAtCols * 128 + (ks % 4) * 32, 16, 1024), idesc, 1);
+        tc::mma_commit(&bars.empty[s]);                    // the centre tiles may be overwritten ...
+        tc::mma_commit(&bars.tfull[b]);                    // ... and the distances read
       }
     }
-    tc::fence_before_sync();
-    __syncthreads();
+  } else {
+    // ---- arg-min sweep: thread = (point row, half of the 128 columns of a tile)
+    const int row = tid & 127, wg = tid >> 7;
+    const uint32_t tlane = tbase + ((uint32_t)((warp & 3) * 32) << 16);
+    float best = INFINITY;
+    int bidx = 0x7fffffff;
+    for (int t = 0; t < NT && ok; ++t) {
+      const int b = t & 1;
+      if (!tc::mbar_wait(&bars.tfull[b], (t >> 1) & 1)) { ok = false; break; }
+      tc::fence_after_sync();
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        float v[32];
+        tc::tmem_ld32(tlane + b * kAtCols + wg * 64 + 32 * q, v);
+        const int c0 = t * kAtCols + wg * 64 + 32 * q;
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+          const float dist = fmaf(-2.f, v[k], cn[c0 + k]);
+          if (dist < best) { best = dist; bidx = c0 + k; }     // ascending index: ties keep the lower
+        }
+      }
+      tc::fence_before_sync();
+      tc::mbar_arrive(&bars.tempty[b]);
+    }
+    // the two column halves of a row meet: lower distance wins, the lower index on a tie
+    if (wg == 1) { best_s[row] = best; idx_s[row] = bidx; }
+    tc::named_bar_sync(1, kAtEpi);
+    if (wg == 0 && ok) {
+      const float ob = best_s[row];
+      const int oi = idx_s[row];
+      if (ob < best || (ob == best && oi < bidx)) bidx = oi;
+      if (row0 + row < N) assign[(size_t)prob * N + row0 + row] = bidx;
+    }
   }
-  if (ok && row0 + tid < N) assign[(size_t)prob * N + row0 + tid] = bidx;
+  if (!ok) atomicExch(status, 6);
   tc::fence_before_sync();
   __syncthreads();
-  if (warp == 0) tc::tmem_dealloc(tbase, kAtCols);
-  if (!ok && tid == 0) atomicExch(status, 6);
+  if (warp == 0) tc::tmem_dealloc(tbase, 2 * kAtCols);
 }
+
+int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
 
 int assign_tc(const void* X, int problems, int N, int D, int C, const float* centres, const float* cnorm, void* chi,
               void* clo, int32_t* assign, int* status, cudaStream_t st) {
@@ -114,15 +146,22 @@ int assign_tc(const void* X, int problems, int N, int D, int C, const float* cen
   prof_mark("k_split_centres", st);
   k_split_centres<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(centres, n, (bf16*)chi, (bf16*)clo);
   MUSE_LAUNCH_OK();
-  const size_t smem = (size_t)(kAtRows + 2 * kAtCols) * D * 2 + 1024;
+  CUtensorMap tx, thi, tlo;
+  int rc = make_tmap_bf16_rows(&tx, X, (uint64_t)problems * N, (uint32_t)D, kAtRows);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&thi, chi, (uint64_t)problems * C, (uint32_t)D, kAtCols);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tlo, clo, (uint64_t)problems * C, (uint32_t)D, kAtCols);
+  if (rc != MUSE_OK) return rc;
+  const int NT = (C + kAtCols - 1) / kAtCols;
+  const int ns = D == 128 ? 2 : 4;                          // ring stages of 64 KB / 32 KB
+  const size_t smem = (size_t)kAtRows * D * 2 + (size_t)ns * 2 * kAtCols * D * 2 + (size_t)NT * kAtCols * 4 + 1024;
   dim3 grid(cdiv(N, kAtRows), problems);
   prof_mark("k_assign_tc", st);
   if (D == 128) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_assign_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_assign_tc<128><<<grid, 128, smem, st>>>((const bf16*)X, N, C, (const bf16*)chi, (const bf16*)clo, cnorm, assign, status);
+    k_assign_tc<128><<<grid, kAtThreads, smem, st>>>(tx, thi, tlo, N, C, ns, cnorm, assign, status);
   } else {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_assign_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_assign_tc<64><<<grid, 128, smem, st>>>((const bf16*)X, N, C, (const bf16*)chi, (const bf16*)clo, cnorm, assign, status);
+    k_assign_tc<64><<<grid, kAtThreads, smem, st>>>(tx, thi, tlo, N, C, ns, cnorm, assign, status);
   }
   MUSE_LAUNCH_OK();
   return MUSE_OK;
