@@ -595,6 +595,7 @@ k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
 // dK and dV leave with plain coalesced read-modify-writes (thread = output dim).
 // ================================================================================================
 constexpr int kFusedThreads = 256, kFusedChunks = 2;
+constexpr int kFusedSplit = 4, kFusedTilesPerCta = 16;    // a cluster with many pair tiles is shared by up to 4 CTAs
 
 struct FusedSmem {
   static constexpr int D = 128;
@@ -616,16 +617,18 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   __shared__ uint32_t tbase_s;
   __shared__ int32_t pid_s[3][kBM];                        // pair ids of the previous, the current and the next tile
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = tid & 127, wg = tid >> 7;
-  const int j = blockIdx.x, pq = blockIdx.y;
+  const int j = blockIdx.x, sub = blockIdx.y, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
   const int32_t* go = goff + (size_t)pq * (nkeys + 1) + j;                // group of plane pl: go[pl * Ck], go[pl * Ck + 1]
   const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const int k0 = ok[0], kall = ok[dm.SB];
-  // any retrieving pair at all?
-  bool any_pair = false;
-  for (int pl = 0; pl < dm.SB; ++pl) any_pair |= go[(size_t)pl * dm.Ck + 1] > go[(size_t)pl * dm.Ck];
-  if (!any_pair) return;
+  int ntiles_all = 0;
+  for (int pl = 0; pl < dm.SB; ++pl) ntiles_all += (go[(size_t)pl * dm.Ck + 1] - go[(size_t)pl * dm.Ck] + kBM - 1) / kBM;
+  // the tiles of the cluster are dealt round-robin to nsub CTAs (one for all but the most retrieved clusters);
+  // CTAs that share a cluster add their dK, dV with atomics
+  const int nsub = min(kFusedSplit, max(1, ntiles_all / kFusedTilesPerCta));
+  if (ntiles_all == 0 || sub >= nsub) return;
   BwdCtx c;
   bwd_setup(c, sm_raw, bar, &tbase_s, SM::cols, tid);
   const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
@@ -651,11 +654,13 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       if (it.pl < dm.SB) { it.t0 = go[(size_t)it.pl * dm.Ck]; it.g1 = go[(size_t)it.pl * dm.Ck + 1]; } else { it.t0 = 0; it.g1 = 0; }
       return it;
     };
-    auto next_of = [&](const Item& a) {
+    auto next1 = [&](const Item& a) {
       if (a.pl >= dm.SB) return a;
       if (a.t0 + kBM < a.g1) { Item it = a; it.t0 += kBM; return it; }
       return first_from(a.pl + 1);
     };
+    auto skip = [&](Item a, int n) { for (int k = 0; k < n; ++k) a = next1(a); return a; };
+    auto next_of = [&](const Item& a) { return skip(a, nsub); };         // this CTA's next tile
     // key / value chunks of this sweep
     __syncthreads();
     const int nkc = min(KC, kall - kc0);                    // keys of the sweep that any plane sees
@@ -681,7 +686,7 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       Lreg = row < nq ? LSE[tt] * kLog2e : 0.f;
       dreg = row < nq ? delta[tt] : 0.f;
     };
-    Item cur = first_from(0), nxt = next_of(cur), nn = next_of(nxt);
+    Item cur = skip(first_from(0), sub), nxt = next_of(cur), nn = next_of(nxt);
     load_pids(cur);
     if (tid < kBM) pid_s[0][tid] = pidreg;
     load_pids(nxt);
@@ -853,8 +858,12 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
         tc::tmem_ld32(tl + (wg == 0 ? SM::cDV : SM::cDK) + ch * kBN + u0, v);
         if (c.ok) {
 #pragma unroll
-          for (int u = 0; u < 32; ++u)
-            if (u0 + u < n) dst[(size_t)(u0 + u) * D] += v[u] * f;
+          for (int u = 0; u < 32; ++u) {
+            if (u0 + u < n) {
+              if (nsub > 1) atomicAdd(dst + (size_t)(u0 + u) * D, v[u] * f);
+              else dst[(size_t)(u0 + u) * D] += v[u] * f;
+            }
+          }
         }
       }
     }
@@ -900,7 +909,7 @@ int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, con
   if (d.D == 128 && getenv("MUSE_RET_BWD_SPLIT") == nullptr) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_bwd_fused_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, FusedSmem::total));
     prof_mark("k_ret_bwd_fused_tc", st);
-    k_ret_bwd_fused_tc<<<dim3(d.Ck, pq), kFusedThreads, FusedSmem::total, st>>>(d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp, (const bf16*)Vp,
+    k_ret_bwd_fused_tc<<<dim3(d.Ck, kFusedSplit, pq), kFusedThreads, FusedSmem::total, st>>>(d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp, (const bf16*)Vp,
                                                                                LSE, delta, off_k, goff, pairs, (bf16*)dq_part, dK_perm, dV_perm, status);
     MUSE_LAUNCH_OK();
     return MUSE_OK;

@@ -272,6 +272,7 @@ k_ret_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, c
 // than 128 visible keys takes further sweeps, whose partial results are merged into the stored rows by
 // their log-sum-exp weights.
 constexpr int kRcThreads = 256, kRcKeys = 128;
+constexpr int kRcSplit = 4, kRcTilesPerCta = 16;          // a cluster with many pair tiles is shared by up to 4 CTAs
 
 struct RcSmem {
   static constexpr int D = 128;
@@ -292,15 +293,17 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   __shared__ int32_t pid_s[3][kTcM];                       // pair ids of the previous, the current and the next tile
   __shared__ float mx_s[2][kTcM], sum_s[2][kTcM], wold_s[kTcM], wnew_s[kTcM];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = tid & 127, wg = tid >> 7;
-  const int j = blockIdx.x, pq = blockIdx.y;
+  const int j = blockIdx.x, sub = blockIdx.y, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
   const int32_t* go = goff + (size_t)pq * (nkeys + 1) + j;                // group of plane pl: go[pl * Ck], go[pl * Ck + 1]
   const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const int k0 = ok[0], kall = ok[dm.SB];
-  bool any_pair = false;
-  for (int pl = 0; pl < dm.SB; ++pl) any_pair |= go[(size_t)pl * dm.Ck + 1] > go[(size_t)pl * dm.Ck];
-  if (!any_pair) return;
+  int ntiles_all = 0;
+  for (int pl = 0; pl < dm.SB; ++pl) ntiles_all += (go[(size_t)pl * dm.Ck + 1] - go[(size_t)pl * dm.Ck] + kTcM - 1) / kTcM;
+  // the tiles of the cluster are dealt round-robin to nsub CTAs (one for all but the most retrieved clusters)
+  const int nsub = min(kRcSplit, max(1, ntiles_all / kRcTilesPerCta));
+  if (ntiles_all == 0 || sub >= nsub) return;
 
   unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
   if (warp == 0) tc::tmem_alloc(&tbase_s, SM::cols);
@@ -328,11 +331,13 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
     if (it.pl < dm.SB) { it.t0 = go[(size_t)it.pl * dm.Ck]; it.g1 = go[(size_t)it.pl * dm.Ck + 1]; }
     return it;
   };
-  auto next_of = [&](const Item& a) {
+  auto next1 = [&](const Item& a) {
     if (a.pl >= dm.SB) return a;
     if (a.t0 + kTcM < a.g1) { Item it = a; it.t0 += kTcM; return it; }
     return first_from(a.pl + 1);
   };
+  auto skip = [&](Item a, int n) { for (int k = 0; k < n; ++k) a = next1(a); return a; };
+  auto next_of = [&](const Item& a) { return skip(a, nsub); };           // this CTA's next tile
   uint4 qreg[kTcM * (D / 8) / kRcThreads];                 // the next tile's Q rows between their loads and their stores
   int pidreg = 0;
   auto load_pids = [&](const Item& it) {
@@ -426,7 +431,7 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
     }
   }
   tc::fence_async_smem();
-  Item cur = first_from(0), nxt = next_of(cur), nn = next_of(nxt);
+  Item cur = skip(first_from(0), sub), nxt = next_of(cur), nn = next_of(nxt);
   load_pids(cur);
   if (tid < kTcM) pid_s[0][tid] = pidreg;
   load_pids(nxt);
@@ -565,7 +570,7 @@ int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, con
   if (d.D == 128 && getenv("MUSE_RET_FWD_STREAM") == nullptr) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_cluster_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, RcSmem::total));
     prof_mark("k_ret_fwd_cluster_tc", st);
-    k_ret_fwd_cluster_tc<<<dim3(d.Ck, d.B * d.Hq), kRcThreads, RcSmem::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k,
+    k_ret_fwd_cluster_tc<<<dim3(d.Ck, kRcSplit, d.B * d.Hq), kRcThreads, RcSmem::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k,
                                                                                  goff, pairs, (bf16*)o_part, l_part, status);
     MUSE_LAUNCH_OK();
     return MUSE_OK;
