@@ -74,6 +74,8 @@ def work_model(w: wl.Workload):
         "k_ret_bwd": ("tensor", heads * 10.0 * D * N * ret_keys),
         "k_ret_bwd_dkdv_tc": ("tensor", heads * 8.0 * D * N * ret_keys),
         "k_ret_bwd_dq_tc": ("tensor", heads * 6.0 * D * N * ret_keys),
+        "k_ret_fwd_cluster_tc": ("tensor", heads * 4.0 * D * N * ret_keys),
+        "k_ret_bwd_fused_tc": ("tensor", heads * 10.0 * D * N * ret_keys),    # S, dP, dQ, dK, dV from one gather
         # merges and assembly
         "k_merge": ("hbm", heads * nd * (8 + e) + part + heads * N * m * 4),
         "k_final_dq": ("hbm", heads * nd * (4 + e) + part),
@@ -219,8 +221,9 @@ def workload_config(w, gain):
 # DRAM bytes per (batch, head) problem from the ncu capture of the headline workload cut to one
 # head (dram__bytes_read.sum + dram__bytes_write.sum; the capture's command and figures are in
 # profiles/top_kernels_headline_one_head.md).  Traffic grows in proportion to the problem count.
-NCU_TRAFFIC_PER_HEAD = {"k_summarize_tc": 1.446e9, "k_local_fwd_tc": 0.0535e9, "k_far_fwd_tc": 2.145e9,
-                        "k_ret_bwd_dkdv_tc": 0.0494e9, "k_far_bwd_tc": 2.374e9, "k_summ_bwd_tc": 1.165e9}
+NCU_TRAFFIC_PER_HEAD = {"k_summarize_tc": 1.430e9, "k_local_fwd_tc": 0.054e9, "k_far_fwd_tc": 1.683e9,
+                        "k_ret_bwd_fused_tc": 0.542e9, "k_ret_fwd_cluster_tc": 0.497e9, "k_far_bwd_tc": 2.374e9,
+                        "k_summ_bwd_tc": 1.146e9}
 
 
 def main():
