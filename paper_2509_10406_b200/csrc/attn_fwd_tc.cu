@@ -166,16 +166,27 @@ __device__ __forceinline__ void tc_teardown(TcCtx& c, int tid, int* status) {
 }
 
 // ---- local (block-diagonal) attention ------------------------------------------------------------
+// 256 threads: thread (row, warpgroup w) owns key columns [32 w, 32 w + 32) of every 64-key tile and
+// output dims [D/2 w, D/2 w + D/2) of its row; the two halves of a row share the running maximum
+// through shared memory.  The next K / V tile is loaded into registers while the current one is on
+// the tensor core.
+constexpr int kLfThreads = 256;
+
 template <int D>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kLfThreads, 2)
 k_local_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ K, const bf16* __restrict__ V,
                float* __restrict__ o_loc, float* __restrict__ lse_loc, int* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar[2];
   __shared__ uint32_t tbase_s;
-  const int tid = threadIdx.x;
-  TcCtx c;
-  tc_setup<D>(c, sm_raw, bar, &tbase_s, tid);
+  __shared__ float mx_s[2][kTcM];
+  constexpr int NKV = kTcN * (D / 8) / kLfThreads;         // 16-byte chunks of a K (or V) tile per thread
+  constexpr int HD = D / 2;
+  const int tid = threadIdx.x, warp = tid >> 5, row = tid & 127, wg = tid >> 7;
+  unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
+  unsigned char *Qs = sm, *Ks = Qs + FwdTcSmem<D>::q_bytes, *Vs = Ks + FwdTcSmem<D>::k_bytes, *Ps = Vs + FwdTcSmem<D>::v_bytes;
+  if (warp == 0) tc::tmem_alloc(&tbase_s, D == 128 ? 256 : 128);
+  if (tid == 0) { tc::mbar_init(&bar[0], 1); tc::mbar_init(&bar[1], 1); tc::mbar_init_fence(); }
   const int tpb = cdiv(dm.Bs, kTcM);
   // heaviest tiles (latest in a block) first
   const int lin = blockIdx.x, qt = tpb - 1 - lin / dm.S, blk = lin % dm.S, pq = blockIdx.y;
@@ -185,21 +196,132 @@ k_local_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ K, 
   const bf16* Qb = Q + (size_t)pq * dm.N * D;
   const bf16* Kb = K + (size_t)pk * dm.N * D;
   const bf16* Vb = V + (size_t)pk * dm.N * D;
-  fill_kmajor<D, kTcM>(c.Qs, nq, [&](int r) { return Qb + (size_t)(q0 + r) * D; }, tid);
-  float o[D], m2 = -INFINITY, l = 0.f;
-#pragma unroll
-  for (int i = 0; i < D; ++i) o[i] = 0.f;
-  const float scale2 = dm.sigma * 1.4426950408889634f;
-  attend_tc<D>(c, Kb, Vb, bstart, q0 + nq, [&](int r) { return q0 + r; }, scale2, o, m2, l, tid);
-  if (c.ok && tid < nq) {
-    const size_t t = (size_t)pq * dm.N + q0 + tid;
-    const float inv = 1.f / l;
-    float4* dst = reinterpret_cast<float4*>(o_loc + t * D);
-#pragma unroll
-    for (int i = 0; i < D / 4; ++i) dst[i] = make_float4(o[4 * i] * inv, o[4 * i + 1] * inv, o[4 * i + 2] * inv, o[4 * i + 3] * inv);
-    lse_loc[t] = (m2 + log2f(l)) * 0.6931471805599453f;
+  for (int e = tid; e < kTcM * (D / 8); e += kLfThreads) {
+    const int r = e / (D / 8), ck = e % (D / 8);
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (r < nq) v = reinterpret_cast<const uint4*>(Qb + (size_t)(q0 + r) * D)[ck];
+    *reinterpret_cast<uint4*>(Qs + (ck >> 3) * kTcM * 128 + tc::sw128_off(r, ck & 7)) = v;
   }
-  tc_teardown<D>(c, tid, status);
+  const int k_lo = bstart, k_hi = q0 + nq;                  // causal: keys up to the tile's last row
+  uint4 kreg[NKV], vreg[NKV];
+  auto load_kv = [&](int c0) {
+    const int nk = min(kTcN, k_hi - c0);
+#pragma unroll
+    for (int k = 0; k < NKV; ++k) {
+      const int e = tid + kLfThreads * k, r = e / (D / 8), ck = e % (D / 8);
+      kreg[k] = r < nk ? __ldg(reinterpret_cast<const uint4*>(Kb + (size_t)(c0 + r) * D) + ck) : make_uint4(0u, 0u, 0u, 0u);
+      vreg[k] = r < nk ? __ldg(reinterpret_cast<const uint4*>(Vb + (size_t)(c0 + r) * D) + ck) : make_uint4(0u, 0u, 0u, 0u);
+    }
+  };
+  load_kv(k_lo);
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tbase = tbase_s, tl = tbase + ((uint32_t)((warp & 3) * 32) << 16);
+  const uint32_t qa = tc::smem_u32(Qs), ka = tc::smem_u32(Ks), va = tc::smem_u32(Vs), pa = tc::smem_u32(Ps);
+  const float scale2 = dm.sigma * 1.4426950408889634f;
+  const int my_limit = q0 + row;                            // last visible key of this row
+  float o[HD], m2 = -INFINITY, l = 0.f;                     // l: this warpgroup's share of the row sum
+#pragma unroll
+  for (int i = 0; i < HD; ++i) o[i] = 0.f;
+  uint32_t ph0 = 0, ph1 = 0;
+  bool ok = true;
+  for (int c0 = k_lo; c0 < k_hi && ok; c0 += kTcN) {
+    const int nk = min(kTcN, k_hi - c0);
+#pragma unroll
+    for (int k = 0; k < NKV; ++k) {
+      const int e = tid + kLfThreads * k, r = e / (D / 8), ck = e % (D / 8);
+      const uint32_t off = (ck >> 3) * kTcN * 128 + tc::sw128_off(r, ck & 7);
+      *reinterpret_cast<uint4*>(Ks + off) = kreg[k];
+      *reinterpret_cast<uint4*>(Vs + off) = vreg[k];
+    }
+    tc::fence_async_smem();
+    tc::fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {
+      tc::fence_after_sync();
+      const uint32_t idesc = tc::idesc_bf16(kTcM, kTcN, 0, 0);
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks)
+        tc::mma_bf16_ss(tbase, tc::smem_desc_sw128(qa + (ks / 4) * kTcM * 128 + (ks % 4) * 32, 16, 1024),
+                        tc::smem_desc_sw128(ka + (ks / 4) * kTcN * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
+      tc::mma_commit(&bar[0]);
+    }
+    __syncwarp();
+    if (c0 + kTcN < k_hi) load_kv(c0 + kTcN);               // next tile: loads fly during the products and the softmax
+    if (!tc::mbar_wait(&bar[0], ph0)) { ok = false; break; }
+    ph0 ^= 1;
+    tc::fence_after_sync();
+    float s[32];
+    tc::tmem_ld32(tl + 32 * wg, s);
+    const int vis = min(nk, my_limit - c0 + 1) - 32 * wg;  // visible columns among this thread's 32
+    float mx = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 32; ++i) { s[i] = i < vis ? s[i] * scale2 : -INFINITY; mx = fmaxf(mx, s[i]); }
+    mx_s[wg][row] = mx;
+    __syncthreads();
+    const float mn = fmaxf(m2, fmaxf(mx_s[0][row], mx_s[1][row]));
+    const float base = mn == -INFINITY ? 0.f : mn;
+    const float resc = tc::fast_exp2(m2 - base);
+    float rs = 0.f;
+    uint32_t pk[16];
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+      __nv_bfloat162 b = __floats2bfloat162_rn(tc::fast_exp2(s[i] - base), tc::fast_exp2(s[i + 1] - base));
+      rs += __low2float(b) + __high2float(b);               // the rounded values, as the P V product sees them
+      pk[i / 2] = *reinterpret_cast<uint32_t*>(&b);
+    }
+    l = l * resc + rs;
+    m2 = mn;
+#pragma unroll
+    for (int ch = 0; ch < 4; ++ch)
+      *reinterpret_cast<uint4*>(Ps + tc::sw128_off(row, 4 * wg + ch)) = make_uint4(pk[ch * 4], pk[ch * 4 + 1], pk[ch * 4 + 2], pk[ch * 4 + 3]);
+    tc::fence_async_smem();
+    tc::fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {
+      tc::fence_after_sync();
+      const uint32_t idesc = tc::idesc_bf16(kTcM, D, 0, 1);
+#pragma unroll
+      for (int ks = 0; ks < kTcN / 16; ++ks)
+        tc::mma_bf16_ss(tbase + kTcN, tc::smem_desc_sw128(pa + ks * 32, 16, 1024),
+                        tc::smem_desc_sw128(va + ks * 16 * 128, kTcN * 128, 1024), idesc, ks > 0);
+      tc::mma_commit(&bar[1]);
+    }
+    __syncwarp();
+    if (resc != 1.f) {
+#pragma unroll
+      for (int i = 0; i < HD; ++i) o[i] *= resc;
+    }
+    if (!tc::mbar_wait(&bar[1], ph1)) { ok = false; break; }
+    ph1 ^= 1;
+    tc::fence_after_sync();
+#pragma unroll
+    for (int d0 = 0; d0 < HD; d0 += 32) {
+      float v[32];
+      tc::tmem_ld32(tl + kTcN + wg * HD + d0, v);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) o[d0 + i] += v[i];
+    }
+    tc::fence_before_sync();
+  }
+  // the two halves of the row sum meet
+  __syncthreads();
+  mx_s[wg][row] = l;
+  __syncthreads();
+  const float lt = mx_s[0][row] + mx_s[1][row];
+  if (ok && row < nq) {
+    const size_t t = (size_t)pq * dm.N + q0 + row;
+    const float inv = 1.f / lt;
+    float4* dst = reinterpret_cast<float4*>(o_loc + t * D + wg * HD);
+#pragma unroll
+    for (int i = 0; i < HD / 4; ++i) dst[i] = make_float4(o[4 * i] * inv, o[4 * i + 1] * inv, o[4 * i + 2] * inv, o[4 * i + 3] * inv);
+    if (wg == 0) lse_loc[t] = (m2 + log2f(lt)) * 0.6931471805599453f;
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tbase, D == 128 ? 256 : 128);
+  if (!ok && tid == 0) atomicExch(status, 1);
 }
 
 // ---- exact retrieval ---------------------------------------------------------------------------------
@@ -554,10 +676,10 @@ int local_fwd_tc(const Dims& d, const void* Q, const void* K, const void* V, flo
   prof_mark("k_local_fwd_tc", st);
   if (d.D == 128) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_local_fwd_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdTcSmem<128>::total));
-    k_local_fwd_tc<128><<<grid, 128, FwdTcSmem<128>::total, st>>>(d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, o_loc, lse_loc, status);
+    k_local_fwd_tc<128><<<grid, kLfThreads, FwdTcSmem<128>::total, st>>>(d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, o_loc, lse_loc, status);
   } else {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_local_fwd_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdTcSmem<64>::total));
-    k_local_fwd_tc<64><<<grid, 128, FwdTcSmem<64>::total, st>>>(d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, o_loc, lse_loc, status);
+    k_local_fwd_tc<64><<<grid, kLfThreads, FwdTcSmem<64>::total, st>>>(d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, o_loc, lse_loc, status);
   }
   MUSE_LAUNCH_OK();
   return MUSE_OK;
