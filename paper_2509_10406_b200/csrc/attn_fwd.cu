@@ -471,24 +471,46 @@ __global__ void k_merge(Dims dm, const float* __restrict__ o_far, const float* _
   const float wf = lf == -INFINITY ? 0.f : expf(lf - mx), wl = ll == -INFINITY ? 0.f : expf(ll - mx);
   tot += wf + wl;
   const float inv = 1.f / tot;
-  float acc[D / 32];
+  // lane owns EPL consecutive output dims: one vector load per input row and lane
+  constexpr int EPL = D / 32;
+  const int dd = lane * EPL;
+  float acc[EPL];
 #pragma unroll
-  for (int k = 0; k < D / 32; ++k) {
-    const int dd = lane + 32 * k;
-    float v = 0.f;
-    if (wf > 0.f) v += wf * o_far[row * D + dd];
-    if (wl > 0.f) v += wl * o_loc[row * D + dd];
-    acc[k] = v;
+  for (int k = 0; k < EPL; ++k) acc[k] = 0.f;
+  if (wf > 0.f) {
+    float x[EPL];
+    ldv<EPL>(o_far + row * D + dd, x);
+#pragma unroll
+    for (int k = 0; k < EPL; ++k) acc[k] = fmaf(wf, x[k], acc[k]);
   }
-  for (int s = 0; s < m; ++s) {
-    const float lp = __shfl_sync(0xffffffffu, lp_mine[s >> 5], s & 31);
-    if (lp == -INFINITY) continue;
-    const float w = expf(lp - mx);
+  if (wl > 0.f) {
+    float x[EPL];
+    ldv<EPL>(o_loc + row * D + dd, x);
 #pragma unroll
-    for (int k = 0; k < D / 32; ++k) acc[k] = fmaf(w, to_f(o_part[(row * m + s) * D + lane + 32 * k]), acc[k]);
+    for (int k = 0; k < EPL; ++k) acc[k] = fmaf(wl, x[k], acc[k]);
+  }
+  // retrieved slots four at a time, so that four independent row loads are in flight
+  for (int s0 = 0; s0 < m; s0 += 4) {
+    float w[4], x[4][EPL];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int s = s0 + u;
+      const float lp = s < m ? __shfl_sync(0xffffffffu, lp_mine[s >> 5], s & 31) : -INFINITY;
+      w[u] = lp == -INFINITY ? 0.f : expf(lp - mx);
+      if (w[u] > 0.f) ldv<EPL>(o_part + (row * m + s) * D + dd, x[u]);
+      else {
+#pragma unroll
+        for (int k = 0; k < EPL; ++k) x[u][k] = 0.f;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int k = 0; k < EPL; ++k) acc[k] = fmaf(w[u], x[u][k], acc[k]);
   }
 #pragma unroll
-  for (int k = 0; k < D / 32; ++k) O[row * D + lane + 32 * k] = from_f<T>(acc[k] * inv);
+  for (int k = 0; k < EPL; ++k) acc[k] *= inv;
+  stv<EPL>(O + row * D + dd, acc);
   if (lane == 0) LSE[row] = mx + logf(tot);
 }
 

@@ -68,6 +68,24 @@ __device__ __forceinline__ void st4(__nv_bfloat16* p, float4 v) {
   *reinterpret_cast<uint2*>(p) = u;
 }
 
+// EPL (2 or 4) consecutive elements as floats / back, one vector access
+template <int EPL> __device__ __forceinline__ void ldv(const float* p, float (&x)[EPL]) {
+  if (EPL == 4) { const float4 v = *reinterpret_cast<const float4*>(p); x[0] = v.x; x[1] = v.y; x[EPL - 2] = v.z; x[EPL - 1] = v.w; }
+  else { const float2 v = *reinterpret_cast<const float2*>(p); x[0] = v.x; x[1] = v.y; }
+}
+template <int EPL> __device__ __forceinline__ void ldv(const __nv_bfloat16* p, float (&x)[EPL]) {
+  if (EPL == 4) { const float4 v = ld4(p); x[0] = v.x; x[1] = v.y; x[EPL - 2] = v.z; x[EPL - 1] = v.w; }
+  else { const uint32_t u = *reinterpret_cast<const uint32_t*>(p); x[0] = __uint_as_float(u << 16); x[1] = __uint_as_float(u & 0xffff0000u); }
+}
+template <int EPL> __device__ __forceinline__ void stv(float* p, const float (&x)[EPL]) {
+  if (EPL == 4) *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[EPL - 2], x[EPL - 1]);
+  else *reinterpret_cast<float2*>(p) = make_float2(x[0], x[1]);
+}
+template <int EPL> __device__ __forceinline__ void stv(__nv_bfloat16* p, const float (&x)[EPL]) {
+  if (EPL == 4) st4(p, make_float4(x[0], x[1], x[EPL - 2], x[EPL - 1]));
+  else { __nv_bfloat162 b = __floats2bfloat162_rn(x[0], x[1]); *reinterpret_cast<uint32_t*>(p) = *reinterpret_cast<uint32_t*>(&b); }
+}
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
