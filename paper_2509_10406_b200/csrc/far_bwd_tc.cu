@@ -5,11 +5,14 @@
 //   S^T   = (kappa_hi + kappa_lo) Q^T,  dPnu^T = nu dO^T                      (tcgen05, TMA-fed tiles)
 //   p     = exp(sigma S + beta - L) on the far set,  g = p (dPnu - delta)      (one thread per cluster)
 //   dnu  += p dO,   dkappa_raw += g Q,   dq^T += kappa^T g                     (tcgen05)
-//   dkappa = sigma (dkappa_raw - (sum_r g) qbar_i),   dS = sum_r g - dkappa.kappa - dnu.nu
+//   dkappa = sigma (dkappa_raw - (sum_r g) qbar_i)
+//   dS = sum_r g - dkappa.kappa - dnu.nu = sum_r g (1 + mu - score) - sum_r p dPnu   (no row dot products)
 // dkappa and dnu are stored as bf16 rows for the key-side pass, dS as fp32.
 #include <cuda.h>
 #include "common.cuh"
 #include "tc05.cuh"
+
+#include <cstdlib>
 
 namespace muse {
 
@@ -42,14 +45,14 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
              const __grid_constant__ CUtensorMap tm_gnu, const bf16* __restrict__ Q, const bf16* __restrict__ dO,
              const float* __restrict__ qbar, const float* __restrict__ LSE, const float* __restrict__ delta,
              const int32_t* __restrict__ off_q, const int32_t* __restrict__ perm_q, const int32_t* __restrict__ sel,
-             const float* __restrict__ beta, float* __restrict__ dQacc, bf16* __restrict__ dkappa,
+             const float* __restrict__ beta, const float* __restrict__ mu, float* __restrict__ dQacc, bf16* __restrict__ dkappa,
              bf16* __restrict__ dnu, float* __restrict__ dS, int grad_by_key_cluster, int* __restrict__ status) {
   using namespace fb;
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar_full, bar1, bar2;
   __shared__ uint32_t tbase_s;
   __shared__ int32_t rows[NP * NR];
-  __shared__ __align__(16) float Ls[NP * NR], ds[NP * NR], qb[D], part[2][TJ], dots[2][TJ];
+  __shared__ __align__(16) float Ls[NP * NR], ds[NP * NR], qb[D], part[2][TJ], dsid[2][TJ];
   const int i = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z;
   const int blk = dm.causal ? pl + 1 : 0, Ck = dm.Ck, NJ = Ck / TJ, MW = Ck >> 5, m = dm.m;
   const int tid = threadIdx.x, warp = tid >> 5, wg = tid >> 7, L = tid & 127;
@@ -130,7 +133,8 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       const float bj = bnext;                               // loaded one tile ahead
       const float sig2 = dm.sigma * kLog2e, bj2 = bj * kLog2e;
       if (jt + 1 < NJ) bnext = beta[ent0 + j + TJ];
-      float gsum = 0.f;
+      float gsum = 0.f, dsum = 0.f;
+      const float mu1 = 1.f + mu[ent0 + j];                               // 1 + accumulated log-mass of cluster j
       for (int p = 0; p < np && ok; ++p) {
         const uint32_t aQ = tc::smem_u32(sm + oQ + p * kRows), aDO = tc::smem_u32(sm + oDO + p * kRows);
         if (tid == 0) {
@@ -185,10 +189,15 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
               const bool far = alive && rb + c + h < ns && !((mk[c + h] >> (j & 31)) & 1u);
-              const float e = fast_exp2(fmaf(s[c + h], sig2, bj2) - Lc[c + h]);
+              const float t2 = fmaf(s[c + h], sig2, bj2);                 // Eq. 6 score in log2 units
+              const float e = fast_exp2(t2 - Lc[c + h]);
               pv[h] = far ? e : 0.f;
               gv[h] = pv[h] * (dp[c + h] - dc[c + h]);
               gsum += gv[h];
+              // dS = sum_r g (1 + mu - score) - sum_r p (dO.nu): the same quantity as
+              // sum_r g - dkappa.kappa - dnu.nu, without the two row dot products
+              dsum = fmaf(gv[h], far ? fmaf(-t2, 0.6931471805599453f, mu1) : 0.f, dsum);    // (an empty cluster has mu = -inf)
+              dsum = fmaf(-pv[h], dp[c + h], dsum);
             }
             __nv_bfloat162 a = __floats2bfloat162_rn(pv[0], pv[1]), b = __floats2bfloat162_rn(gv[0], gv[1]);
             pw[c >> 1] = *reinterpret_cast<uint32_t*>(&a);
@@ -242,52 +251,37 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #endif
       // ---- tile read-out: warpgroup 0 -> dnu, warpgroup 1 -> dkappa; both need sum_r g
       part[wg][L] = gsum;
+      dsid[wg][L] = dsum;
       __syncthreads();
       const float gtot = part[0][L] + part[1][L];
-      float dot = 0.f;
       // gradient entry: [plane][i][j] like the summaries, or [plane][j][i] so that the key-side
       // pass finds the 128 query clusters of one key cluster in one contiguous tile
       const size_t gent = grad_by_key_cluster ? (((size_t)pq * dm.SB + pl) * Ck + j) * dm.Cq + i : ent0 + j;
-      bf16* dst = (wg == 0 ? dnu : dkappa) + gent * D;
 #pragma unroll
       for (int d0 = 0; d0 < D; d0 += 32) {
         float v[32];
         tc::tmem_ld32(tlane + (wg == 0 ? cDNU : cDKA) + d0, v);
-        // operands of this 32-wide slice first (vector loads), arithmetic after
-        float qv[32];
-        uint4 ra[4], rb[4];
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-          const int d = d0 + 8 * ch, kb = d >> 6, c = (d & 63) >> 3;
-          const uint32_t off = kb * TJ * 128 + tc::sw128_off(L, c);
-          ra[ch] = *reinterpret_cast<const uint4*>(sm + (wg == 0 ? oNu : oHi) + off);
-          rb[ch] = wg == 0 ? make_uint4(0u, 0u, 0u, 0u) : *reinterpret_cast<const uint4*>(sm + oLo + off);
-          const float4 q0 = *reinterpret_cast<const float4*>(qb + d), q1 = *reinterpret_cast<const float4*>(qb + d + 4);
-          qv[8 * ch] = q0.x; qv[8 * ch + 1] = q0.y; qv[8 * ch + 2] = q0.z; qv[8 * ch + 3] = q0.w;
-          qv[8 * ch + 4] = q1.x; qv[8 * ch + 5] = q1.y; qv[8 * ch + 6] = q1.z; qv[8 * ch + 7] = q1.w;
-        }
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           const int d = d0 + 8 * ch;
           float x[8];
+          if (wg == 0) {
 #pragma unroll
-          for (int e = 0; e < 8; ++e)      // rounded to the stored bf16 value so that dS matches what the key-side pass reads
-            x[e] = __bfloat162float(__float2bfloat16_rn(wg == 0 ? v[8 * ch + e] : dm.sigma * (v[8 * ch + e] - gtot * qv[8 * ch + e])));
-          const bf16* ha = reinterpret_cast<const bf16*>(&ra[ch]);
-          const bf16* hb = reinterpret_cast<const bf16*>(&rb[ch]);
+            for (int e = 0; e < 8; ++e) x[e] = v[8 * ch + e];
+          } else {
+            const float4 q0 = *reinterpret_cast<const float4*>(qb + d), q1 = *reinterpret_cast<const float4*>(qb + d + 4);
+            const float qv[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
 #pragma unroll
-          for (int e = 0; e < 8; ++e) dot = fmaf(x[e], __bfloat162float(ha[e]) + __bfloat162float(hb[e]), dot);
+            for (int e = 0; e < 8; ++e) x[e] = dm.sigma * (v[8 * ch + e] - gtot * qv[e]);
+          }
           uint32_t w[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) { __nv_bfloat162 b2 = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]); w[e] = *reinterpret_cast<uint32_t*>(&b2); }
-          // back into this thread's own row of the (now consumed) nu / kappa_hi tile; the rows leave
-          // through a cooperative, fully coalesced copy below instead of 16-byte scattered stores
+          // into this thread's own row of the (consumed) nu / kappa_hi tile, which then leaves as one TMA box
           const int kb = d >> 6, c = (d & 63) >> 3;
           *reinterpret_cast<uint4*>(sm + (wg == 0 ? oNu : oHi) + kb * TJ * 128 + tc::sw128_off(L, c)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
-      (void)dst;
-      dots[wg][L] = dot;
       // the two gradient tiles leave by TMA: 128 rows of 256 bytes each, Cq entries apart in the
       // [plane][j][i] layout (adjacent in the [plane][i][j] one)
       tc::fence_async_smem();
@@ -300,7 +294,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
         tc::tma_store_commit();
       }
       tc::fence_before_sync();
-      if (wg == 0 && ok) dS[gent] = gtot - dots[0][L] - dots[1][L];
+      if (wg == 0 && ok) dS[gent] = dsid[0][L] + dsid[1][L];
 #ifdef MUSE_PHASE_CLOCKS
       k4_ = clock64();
       pc[0] += k1_ - k0_; pc[1] += k2_ - k1_; pc[2] += k3_ - k2_; pc[3] += k4_ - k3_; pc[4] += 1; pc[5] = np;
@@ -360,7 +354,7 @@ int far_bwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const void* dO,
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_bwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prof_mark("k_far_bwd_tc", st);
   k_far_bwd_tc<<<dim3(d.Cq, d.SB, d.B * d.Hq), fb::THREADS, smem, st>>>(
-      d, khi, klo, nu, gka, gnu, (const bf16*)Q, (const bf16*)dO, qbar, LSE, delta, off_q, perm_q, sel, sp.beta, dQacc, (bf16*)dkappa,
+      d, khi, klo, nu, gka, gnu, (const bf16*)Q, (const bf16*)dO, qbar, LSE, delta, off_q, perm_q, sel, sp.beta, sp.mu, dQacc, (bf16*)dkappa,
       (bf16*)dnu, dS, grad_by_key_cluster, status);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
