@@ -1,7 +1,7 @@
 // Far-field backward on the tensor cores (bf16 mode, D = 128, Ck a multiple of 128, <= 1024).
 // One CTA per (query cluster i, plane, head) segment.  Clusters sit on the MMA M side (128 per
-// tile, one TMEM lane each), the segment's queries on the N side (64 per pass, two passes
-// resident).  Per cluster tile, with L the merged log-sum-exp and delta = dO.O:
+// tile, one TMEM lane each), the segment's queries on the N side (64 per sweep; a longer segment
+// takes further sweeps that add to the stored gradients).  Per cluster tile, with L the merged log-sum-exp and delta = dO.O:
 //   S^T   = (kappa_hi + kappa_lo) Q^T,  dPnu^T = nu dO^T                      (tcgen05, TMA-fed tiles)
 //   p     = exp(sigma S + beta - L) on the far set,  g = p (dPnu - delta)      (one thread per cluster)
 //   dnu  += p dO,   dkappa_raw += g Q,   dq^T += kappa^T g                     (tcgen05)
@@ -22,13 +22,16 @@ int make_tmap_bf16_nd(void* out_map, const void* base, int rank, const uint64_t*
                       const uint32_t* box);
 
 namespace fb {
-constexpr int D = 128, TJ = 128, NR = 64, NP = 2, THREADS = 256;
+constexpr int D = 128, TJ = 128, NR = 64, NP = 1, THREADS = 256;
 constexpr int kTile = TJ * D * 2;                 // 32 KB operand tile [128][128] bf16
 constexpr int kRows = NR * D * 2;                 // 16 KB tile of 64 query rows
 constexpr int oHi = 0, oLo = oHi + kTile, oNu = oLo + kTile;
 constexpr int oQ = oNu + kTile, oDO = oQ + NP * kRows;
 constexpr int oPt = oDO + NP * kRows, oGt = oPt + TJ * NR * 2;
-constexpr int oMask = oGt + TJ * NR * 2;          // [NP*NR rows][Ck/32] words follow
+// gradient rows on their way out: dkappa is staged in the (consumed) P / G tiles, dnu in a tile of its own,
+// so that the three operand tiles are free for the next cluster tile as soon as the MMAs have finished
+constexpr int oStK = oPt, oStN = oGt + TJ * NR * 2;
+constexpr int oMask = oStN + kTile;               // [NP*NR rows][Ck/32] words follow
 constexpr uint32_t cS = 0, cDP = 64, cDNU = 128, cDKA = 256, cDQ = 384;   // TMEM columns
 constexpr float kLog2e = 1.4426950408889634f;
 }  // namespace fb
@@ -111,25 +114,24 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     long long pc[6] = {0, 0, 0, 0, 0, 0};
 #endif
     float bnext = beta[ent0 + L];
+    auto issue_tile = [&](int jt_) {                        // thread 0: the three operand tiles of cluster tile jt_
+      tc::mbar_expect_tx(&bar_full, 3 * kTile);
+      const int row = (int)(ent0 + (size_t)jt_ * TJ);
+      tc::tma_load_2d(sm + oHi, &tm_khi, 0, row, &bar_full); tc::tma_load_2d(sm + oHi + TJ * 128, &tm_khi, 64, row, &bar_full);
+      tc::tma_load_2d(sm + oLo, &tm_klo, 0, row, &bar_full); tc::tma_load_2d(sm + oLo + TJ * 128, &tm_klo, 64, row, &bar_full);
+      tc::tma_load_2d(sm + oNu, &tm_nu, 0, row, &bar_full); tc::tma_load_2d(sm + oNu + TJ * 128, &tm_nu, 64, row, &bar_full);
+    };
+    const bool later_sweep = s0 > p0;                       // gradients of earlier sweeps are already stored: add to them
+    if (tid == 0) {
+      if (later_sweep) tc::tma_store_wait_all();
+      issue_tile(0);
+    }
+    if (later_sweep) __syncthreads();
     for (int jt = 0; jt < NJ && ok; ++jt) {
       const int j = jt * TJ + L;
 #ifdef MUSE_PHASE_CLOCKS
       long long k0_ = clock64(), k1_ = 0, k2_ = 0, k3_ = 0, k4_ = 0;
 #endif
-      if (tid == 0) {
-        tc::tma_store_wait_read();            // the previous tile's gradient stores have read the kappa_hi / nu buffers
-        tc::mbar_expect_tx(&bar_full, 3 * kTile);
-        const int row = (int)(ent0 + (size_t)jt * TJ);
-        tc::tma_load_2d(sm + oHi, &tm_khi, 0, row, &bar_full); tc::tma_load_2d(sm + oHi + TJ * 128, &tm_khi, 64, row, &bar_full);
-        tc::tma_load_2d(sm + oLo, &tm_klo, 0, row, &bar_full); tc::tma_load_2d(sm + oLo + TJ * 128, &tm_klo, 64, row, &bar_full);
-        tc::tma_load_2d(sm + oNu, &tm_nu, 0, row, &bar_full); tc::tma_load_2d(sm + oNu + TJ * 128, &tm_nu, 64, row, &bar_full);
-        if (jt + 1 < NJ) {                    // start pulling the next cluster tile into L2 while this one is processed
-          const int nrow = row + TJ;
-          tc::tma_prefetch_2d(&tm_khi, 0, nrow); tc::tma_prefetch_2d(&tm_khi, 64, nrow);
-          tc::tma_prefetch_2d(&tm_klo, 0, nrow); tc::tma_prefetch_2d(&tm_klo, 64, nrow);
-          tc::tma_prefetch_2d(&tm_nu, 0, nrow); tc::tma_prefetch_2d(&tm_nu, 64, nrow);
-        }
-      }
       const float bj = bnext;                               // loaded one tile ahead
       const float sig2 = dm.sigma * kLog2e, bj2 = bj * kLog2e;
       if (jt + 1 < NJ) bnext = beta[ent0 + j + TJ];
@@ -138,7 +140,10 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       for (int p = 0; p < np && ok; ++p) {
         const uint32_t aQ = tc::smem_u32(sm + oQ + p * kRows), aDO = tc::smem_u32(sm + oDO + p * kRows);
         if (tid == 0) {
-          if (p == 0) { if (!tc::mbar_wait(&bar_full, ph_full)) ok = false; }
+          if (p == 0) {
+            if (!tc::mbar_wait(&bar_full, ph_full)) ok = false;
+            tc::tma_store_wait_read();        // the previous tile's stores have read the P / G tiles, which are written again below
+          }
           tc::fence_after_sync();
           const uint32_t idesc = tc::idesc_bf16(TJ, NR, 0, 0);
 #pragma unroll
@@ -246,6 +251,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
         tc::fence_after_sync();
       }
       ph_full ^= 1;
+      if (tid == 0 && jt + 1 < NJ && ok) issue_tile(jt + 1);    // every MMA on the operand tiles has completed
 #ifdef MUSE_PHASE_CLOCKS
       k3_ = clock64();
 #endif
@@ -277,9 +283,16 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
           uint32_t w[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) { __nv_bfloat162 b2 = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]); w[e] = *reinterpret_cast<uint32_t*>(&b2); }
-          // into this thread's own row of the (consumed) nu / kappa_hi tile, which then leaves as one TMA box
+          // into this thread's own row of the staging tile, which then leaves as one TMA box
           const int kb = d >> 6, c = (d & 63) >> 3;
-          *reinterpret_cast<uint4*>(sm + (wg == 0 ? oNu : oHi) + kb * TJ * 128 + tc::sw128_off(L, c)) = make_uint4(w[0], w[1], w[2], w[3]);
+          if (later_sweep) {
+            const bf16* old = (wg == 0 ? dnu : dkappa) + gent * D + d;
+            const float4 o0 = ld4(old), o1 = ld4(old + 4);
+            x[0] += o0.x; x[1] += o0.y; x[2] += o0.z; x[3] += o0.w; x[4] += o1.x; x[5] += o1.y; x[6] += o1.z; x[7] += o1.w;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { __nv_bfloat162 b2 = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]); w[e] = *reinterpret_cast<uint32_t*>(&b2); }
+          }
+          *reinterpret_cast<uint4*>(sm + (wg == 0 ? oStN : oStK) + kb * TJ * 128 + tc::sw128_off(L, c)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
       // the two gradient tiles leave by TMA: 128 rows of 256 bytes each, Cq entries apart in the
@@ -289,12 +302,12 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       if (tid == 0 && ok) {
         const int c1 = grad_by_key_cluster ? i : 0;
         const int c2 = grad_by_key_cluster ? (pq * dm.SB + pl) * Ck + jt * TJ : (int)(ent0 + (size_t)jt * TJ);
-        tc::tma_store_3d(&tm_gnu, sm + oNu, 0, c1, c2); tc::tma_store_3d(&tm_gnu, sm + oNu + TJ * 128, 64, c1, c2);
-        tc::tma_store_3d(&tm_gka, sm + oHi, 0, c1, c2); tc::tma_store_3d(&tm_gka, sm + oHi + TJ * 128, 64, c1, c2);
+        tc::tma_store_3d(&tm_gnu, sm + oStN, 0, c1, c2); tc::tma_store_3d(&tm_gnu, sm + oStN + TJ * 128, 64, c1, c2);
+        tc::tma_store_3d(&tm_gka, sm + oStK, 0, c1, c2); tc::tma_store_3d(&tm_gka, sm + oStK + TJ * 128, 64, c1, c2);
         tc::tma_store_commit();
       }
       tc::fence_before_sync();
-      if (wg == 0 && ok) dS[gent] = dsid[0][L] + dsid[1][L];
+      if (wg == 0 && ok) dS[gent] = (later_sweep ? dS[gent] : 0.f) + dsid[0][L] + dsid[1][L];
 #ifdef MUSE_PHASE_CLOCKS
       k4_ = clock64();
       pc[0] += k1_ - k0_; pc[1] += k2_ - k1_; pc[2] += k3_ - k2_; pc[3] += k4_ - k3_; pc[4] += 1; pc[5] = np;

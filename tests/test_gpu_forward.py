@@ -18,6 +18,10 @@ EDGE = {
     "one_qcluster": CASES["tiny"].with_(Cq=1, N=512),
     "tiny_blocks": CASES["tiny"].with_(N=64, Cq=2, Ck=8, m=8, components=4),
     "ragged_f32_d128": CASES["d128"].with_(dtype="f32", N=1000, Hq=1, Cq=8, Ck=24, m=3),
+    # segments of ~128 queries (several 64-query sweeps per segment in the tensor far-field kernels) and key
+    # clusters of ~128 keys (several key sweeps in the retrieval kernels)
+    "long_segments": CASES["d128"].with_(Hq=1, Hkv=1, N=4096, S=4, Cq=8, Ck=128, m=4),
+    "long_clusters": CASES["d128"].with_(Hq=1, Hkv=1, N=4096, S=4, Cq=16, Ck=16, m=4),
 }
 
 
