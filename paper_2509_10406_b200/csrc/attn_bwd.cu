@@ -646,10 +646,11 @@ int far_bwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const void* dO,
 bool summ_bwd_tc_supported(const Dims& d, int dtype);
 int summ_bwd_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* off_q, const float* qbar,
                 const float* mu, const void* dkappa, const void* dnu, const float* dS, float* dK_perm, float* dV_perm,
-                int* status, cudaStream_t st);
+                void* qsplit, int* status, cudaStream_t st);
 
 struct BwdWs {
   int32_t *status, *off_q, *perm_q, *sort_scratch, *ret_scratch;
+  __nv_bfloat16* qsplit;
   float *delta, *dQacc, *dq_part, *dK_orig, *dV_orig, *dK_perm, *dV_perm, *dkappa, *dnu, *dS;
 };
 
@@ -671,6 +672,7 @@ static BwdWs bwd_ws(const Dims& d, Arena& ar) {
   w.dkappa = ar.take<float>(ent * d.D);
   w.dnu = ar.take<float>(ent * d.D);
   w.dS = ar.take<float>(ent);
+  w.qsplit = ar.take<__nv_bfloat16>(2 * pq * d.Cq * d.D);
   return w;
 }
 
@@ -752,7 +754,7 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
     }
     const size_t ssm = (size_t)(5 * kTile * (D + 4) + kTile * kLDP) * sizeof(float);
     if (summ_tc) {
-      rc = summ_bwd_tc(d, Kp, Vp, off_k, w.off_q, qbar, mu, w.dkappa, w.dnu, w.dS, w.dK_perm, w.dV_perm, w.status, st);
+      rc = summ_bwd_tc(d, Kp, Vp, off_k, w.off_q, qbar, mu, w.dkappa, w.dnu, w.dS, w.dK_perm, w.dV_perm, w.qsplit, w.status, st);
       if (rc != MUSE_OK) return rc;
     } else if (far_tc) {
       typedef __nv_bfloat16 GB;

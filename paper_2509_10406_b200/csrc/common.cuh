@@ -116,6 +116,10 @@ int summarize(const Dims& d, int dtype, const void* K, const void* V, const int3
               cudaStream_t st);
 size_t summarize_ws_bytes(const Dims& d, int dtype);
 
+// sigma * qbar as two bf16 planes (hi + lo keeps ~16 mantissa bits), [B*Hq*Cq][D] each: the tensor-core
+// summary kernels load their centroid tiles from these by TMA instead of converting them per CTA
+int split_qbar(const Dims& d, const float* qbar, void* qhi, void* qlo, cudaStream_t st);
+
 // dipole correction (dipole.cu): construction at summary time, consumption after the far field
 size_t dipole_ws_bytes(const Dims& d, int dtype);
 int dipole_build(const Dims& d, int dtype, const void* Kp, const void* Vp, const int32_t* off_k, const float* mu,

@@ -37,12 +37,13 @@ int make_tmap_bf16_pitched(void* out_map, const void* base, uint64_t rows, uint6
 __global__ void __launch_bounds__(sb::THREADS, 1)
 k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_constant__ CUtensorMap tm_dnu,
               const __grid_constant__ CUtensorMap tm_K, const __grid_constant__ CUtensorMap tm_V,
-              const int32_t* __restrict__ off_k, const int32_t* __restrict__ off_q, const float* __restrict__ qbar,
+              const __grid_constant__ CUtensorMap tm_qhi, const __grid_constant__ CUtensorMap tm_qlo,
+              const int32_t* __restrict__ off_k, const int32_t* __restrict__ off_q,
               const float* __restrict__ mu, const float* __restrict__ dS, float* __restrict__ dK_perm,
               float* __restrict__ dV_perm, int* __restrict__ status) {
   using namespace sb;
   extern __shared__ __align__(1024) unsigned char sm_raw[];
-  __shared__ uint64_t bar_g[2], bar_kv, bar_l, bar1, bar2;
+  __shared__ uint64_t bar_g[2], bar_kv, bar_q, bar_l, bar1, bar2;
   __shared__ uint32_t tbase_s;
   const int j = blockIdx.x, pq = blockIdx.y;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
@@ -54,14 +55,14 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
   unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
   if (warp == 0) tc::tmem_alloc(&tbase_s, 512);
   if (tid == 0) {
-    tc::mbar_init(&bar_g[0], 1); tc::mbar_init(&bar_g[1], 1); tc::mbar_init(&bar_kv, 1); tc::mbar_init(&bar_l, 1);
+    tc::mbar_init(&bar_g[0], 1); tc::mbar_init(&bar_g[1], 1); tc::mbar_init(&bar_kv, 1); tc::mbar_init(&bar_q, 1); tc::mbar_init(&bar_l, 1);
     tc::mbar_init(&bar1, 1); tc::mbar_init(&bar2, 1); tc::mbar_init_fence();
   }
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
   const uint32_t tbase = tbase_s, tlane = tbase + ((uint32_t)((warp & 3) * 32) << 16);
-  uint32_t ph_g[2] = {0, 0}, ph_kv = 0, ph_l = 0, ph1 = 0, ph2 = 0;
+  uint32_t ph_g[2] = {0, 0}, ph_kv = 0, ph_q = 0, ph_l = 0, ph1 = 0, ph2 = 0;
   bool ok = true;
   const uint32_t aQhi = tc::smem_u32(sm + oQhi), aQlo = tc::smem_u32(sm + oQlo), aK = tc::smem_u32(sm + oK),
                  aV = tc::smem_u32(sm + oV), aW = tc::smem_u32(sm + oW), aWc = tc::smem_u32(sm + oWc);
@@ -101,28 +102,13 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
       };
       PCLK(7)
       __syncthreads();                                    // every MMA that read the centroid tiles has completed (bar2 waited)
-      if (tid == 0 && pl0 < dm.SB) issue_grad(pl0, 0);
-      // sigma * qbar tile as bf16 hi + lo (thread = row, warpgroup = half of the 16-byte chunks)
-      {
-        const float* src = qbar + ((size_t)pq * dm.Cq + ic) * D;
-#pragma unroll
-        for (int c8 = 0; c8 < D / 16; ++c8) {
-          const int ck = wg * (D / 16) + c8;
-          uint32_t wh[4], wl[4];
-          const float4 f0 = in_range ? ld4(src + ck * 8) : make_float4(0.f, 0.f, 0.f, 0.f);
-          const float4 f1 = in_range ? ld4(src + ck * 8 + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-          const float x[8] = {f0.x * dm.sigma, f0.y * dm.sigma, f0.z * dm.sigma, f0.w * dm.sigma,
-                              f1.x * dm.sigma, f1.y * dm.sigma, f1.z * dm.sigma, f1.w * dm.sigma};
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            __nv_bfloat162 hh = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]);
-            __nv_bfloat162 ll = __floats2bfloat162_rn(x[2 * e] - __low2float(hh), x[2 * e + 1] - __high2float(hh));
-            wh[e] = *reinterpret_cast<uint32_t*>(&hh); wl[e] = *reinterpret_cast<uint32_t*>(&ll);
-          }
-          const uint32_t off = (ck >> 3) * TI * 128 + tc::sw128_off(L, ck & 7);
-          *reinterpret_cast<uint4*>(sm + oQhi + off) = make_uint4(wh[0], wh[1], wh[2], wh[3]);
-          *reinterpret_cast<uint4*>(sm + oQlo + off) = make_uint4(wl[0], wl[1], wl[2], wl[3]);
-        }
+      if (tid == 0) {
+        // sigma * qbar tile as bf16 hi + lo operands (split once per layer), and the first gradient tiles
+        tc::mbar_expect_tx(&bar_q, 2 * kTile);
+        const int r = pq * dm.Cq + i0;
+        tc::tma_load_2d(sm + oQhi, &tm_qhi, 0, r, &bar_q); tc::tma_load_2d(sm + oQhi + TI * 128, &tm_qhi, 64, r, &bar_q);
+        tc::tma_load_2d(sm + oQlo, &tm_qlo, 0, r, &bar_q); tc::tma_load_2d(sm + oQlo + TI * 128, &tm_qlo, 64, r, &bar_q);
+        if (pl0 < dm.SB) issue_grad(pl0, 0);
       }
       // which planes hold a non-empty segment of query cluster i (others were never written by the far-field pass)
       uint32_t livemask = 0u;
@@ -130,11 +116,9 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         const int blk = dm.causal ? pl + 1 : 0;
         if (in_range && oq[(size_t)blk * dm.Cq + i + 1] > oq[(size_t)blk * dm.Cq + i]) livemask |= 1u << pl;
       }
-      tc::fence_async_smem();
-      tc::fence_before_sync();
-      __syncthreads();
       // tilt logits l_iu = sigma qbar_i . k_u, the same for every plane: once per centroid tile
       if (tid == 0) {
+        if (!tc::mbar_wait(&bar_q, ph_q)) ok = false;
         tc::fence_after_sync();
         const uint32_t idesc = tc::idesc_bf16(TI, NU, 0, 0);
 #pragma unroll
@@ -147,6 +131,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
                           tc::smem_desc_sw128(aK + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, 1);
         tc::mma_commit(&bar_l);
       }
+      ph_q ^= 1;
       __syncwarp();
       if (!tc::mbar_wait(&bar_l, ph_l)) ok = false;       // from here on the low tile's space is free
       ph_l ^= 1;
@@ -299,7 +284,16 @@ int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t
 
 int summ_bwd_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* off_q, const float* qbar,
                 const float* mu, const void* dkappa, const void* dnu, const float* dS, float* dK_perm, float* dV_perm,
-                int* status, cudaStream_t st) {
+                void* qsplit, int* status, cudaStream_t st) {
+  // qsplit: 2 * B*Hq*Cq*D bf16 of scratch for the split centroids
+  bf16* qhi = (bf16*)qsplit;
+  bf16* qlo = qhi + (size_t)d.B * d.Hq * d.Cq * sb::D;
+  int rcq = split_qbar(d, qbar, qhi, qlo, st);
+  if (rcq != MUSE_OK) return rcq;
+  CUtensorMap tqh, tql;
+  rcq = make_tmap_bf16_rows(&tqh, qhi, (uint64_t)d.B * d.Hq * d.Cq, sb::D, sb::TI);
+  if (rcq == MUSE_OK) rcq = make_tmap_bf16_rows(&tql, qlo, (uint64_t)d.B * d.Hq * d.Cq, sb::D, sb::TI);
+  if (rcq != MUSE_OK) return rcq;
   CUtensorMap tdka, tdnu, tK, tV;
   const uint64_t grows = (uint64_t)d.B * d.Hq * d.SB * d.Ck * d.Cq;       // gradient entries, [plane][j][i]
   int rc = make_tmap_bf16_rows(&tdka, dkappa, grows, sb::D, sb::TI);
@@ -309,7 +303,7 @@ int summ_bwd_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* of
   if (rc != MUSE_OK) return rc;
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, sb::total));
   prof_mark("k_summ_bwd_tc", st);
-  k_summ_bwd_tc<<<dim3(d.Ck, d.B * d.Hq), sb::THREADS, sb::total, st>>>(d, tdka, tdnu, tK, tV, off_k, off_q, qbar, mu, dS, dK_perm,
+  k_summ_bwd_tc<<<dim3(d.Ck, d.B * d.Hq), sb::THREADS, sb::total, st>>>(d, tdka, tdnu, tK, tV, tqh, tql, off_k, off_q, mu, dS, dK_perm,
                                                                 dV_perm, status);
   MUSE_LAUNCH_OK();
   return MUSE_OK;

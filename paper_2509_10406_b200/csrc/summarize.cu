@@ -9,7 +9,7 @@ namespace muse {
 
 bool summarize_tc_supported(const Dims& d, int dtype);
 int summarize_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const float* qbar, const SummPtrs& sp,
-                 int* status, cudaStream_t stream);
+                 void* qsplit, int* status, cudaStream_t stream);
 
 SummLayout summ_layout(const Dims& d, int dtype) {
   const size_t es = dtype == MUSE_F32 ? 4 : 2;
@@ -170,7 +170,7 @@ k_summarize(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const i
 
 template <class T, int D>
 static int summarize_planes(const Dims& d, int dtype, const T* Kp, const T* Vp, const int32_t* off_k, const float* qbar,
-                            const SummLayout& L, char* base, int32_t* status, cudaStream_t st);
+                            const SummLayout& L, char* base, void* qsplit, int32_t* status, cudaStream_t st);
 
 template <class T, int D>
 static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const int32_t* assign_k,
@@ -194,16 +194,17 @@ static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const i
   Arena ar(ws);
   int32_t* status = ar.take<int32_t>(sort_ws_elems(d.N, d.Ck * d.S) * (size_t)pk + 64) + sort_ws_elems(d.N, d.Ck * d.S) * (size_t)pk;
   MUSE_CUDA_OK(cudaMemsetAsync(status, 0, 64 * sizeof(int32_t), st));     // 64 words after the sort scratch
-  rc = summarize_planes<T, D>(d, dtype, Kp, Vp, off_k, qbar, L, base, status, st);
+  void* qsplit = ar.take<__nv_bfloat16>(2 * (size_t)d.B * d.Hq * d.Cq * d.D);   // split centroids for the tensor kernel
+  rc = summarize_planes<T, D>(d, dtype, Kp, Vp, off_k, qbar, L, base, qsplit, status, st);
   if (rc != MUSE_OK || !d.dipole) return rc;
   return dipole_build(d, dtype, Kp, Vp, off_k, summ_ptrs(L, base).mu, base + L.cbar, (char*)ws + ar.used, status, st);
 }
 
 template <class T, int D>
 static int summarize_planes(const Dims& d, int dtype, const T* Kp, const T* Vp, const int32_t* off_k, const float* qbar,
-                            const SummLayout& L, char* base, int32_t* status, cudaStream_t st) {
+                            const SummLayout& L, char* base, void* qsplit, int32_t* status, cudaStream_t st) {
   if (summarize_tc_supported(d, dtype) && getenv("MUSE_SUMM_FWD_SIMT") == nullptr)
-    return summarize_tc(d, Kp, Vp, off_k, qbar, summ_ptrs(L, base), status, st);
+    return summarize_tc(d, Kp, Vp, off_k, qbar, summ_ptrs(L, base), qsplit, status, st);
   const size_t smem = (size_t)(kSumI * (D + 4) + kSumKC * (2 * D + 4) + kSumI * (kSumKC + 1)) * sizeof(float);
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid(d.Ck, cdiv(d.Cq, kSumI), d.B * d.Hq);
@@ -216,6 +217,7 @@ static int summarize_planes(const Dims& d, int dtype, const T* Kp, const T* Vp, 
 size_t summarize_ws_bytes(const Dims& d, int dtype) {
   Arena ar(nullptr);
   ar.take<int32_t>((size_t)d.B * d.Hkv * sort_ws_elems(d.N, d.Ck * d.S) + 64);
+  ar.take<__nv_bfloat16>(2 * (size_t)d.B * d.Hq * d.Cq * d.D);
   return ar.used + dipole_ws_bytes(d, dtype);
 }
 

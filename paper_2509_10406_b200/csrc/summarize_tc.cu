@@ -30,13 +30,31 @@ constexpr int total = oStage + 3 * kTile + 1024;
 constexpr uint32_t cL = 0, cUk = 64, cUv = 192;
 }  // namespace st
 
+__global__ void k_split_qbar(const float* __restrict__ qbar, long long n, float sigma, bf16* __restrict__ hi, bf16* __restrict__ lo) {
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= n) return;
+  const float x = qbar[e] * sigma;
+  const bf16 h = __float2bfloat16_rn(x);
+  hi[e] = h;
+  lo[e] = __float2bfloat16_rn(x - __bfloat162float(h));
+}
+
+int split_qbar(const Dims& d, const float* qbar, void* qhi, void* qlo, cudaStream_t st) {
+  const long long n = (long long)d.B * d.Hq * d.Cq * d.D;
+  prof_mark("k_split_qbar", st);
+  k_split_qbar<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(qbar, n, d.sigma, (bf16*)qhi, (bf16*)qlo);
+  MUSE_LAUNCH_OK();
+  return MUSE_OK;
+}
+
 __global__ void __launch_bounds__(st::THREADS, 1)
 k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_constant__ CUtensorMap tm_V,
                const __grid_constant__ CUtensorMap tm_okhi, const __grid_constant__ CUtensorMap tm_oklo,
-               const __grid_constant__ CUtensorMap tm_onu, const int32_t* __restrict__ off_k, const float* __restrict__ qbar, SummPtrs sp, int* __restrict__ status) {
+               const __grid_constant__ CUtensorMap tm_onu, const __grid_constant__ CUtensorMap tm_qhi,
+               const __grid_constant__ CUtensorMap tm_qlo, const int32_t* __restrict__ off_k, SummPtrs sp, int* __restrict__ status) {
   using namespace st;
   extern __shared__ __align__(1024) unsigned char sm_raw[];
-  __shared__ uint64_t bar_kv, bar1, bar2;
+  __shared__ uint64_t bar_kv, bar_q, bar1, bar2;
   __shared__ uint32_t tbase_s;
   const int j = blockIdx.x, i0 = blockIdx.y * TI, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
@@ -44,35 +62,22 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
   unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
   const int32_t* off = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   if (warp == 0) tc::tmem_alloc(&tbase_s, 512);
-  if (tid == 0) { tc::mbar_init(&bar_kv, 1); tc::mbar_init(&bar1, 1); tc::mbar_init(&bar2, 1); tc::mbar_init_fence(); }
-  // sigma * qbar rows as bf16 hi (warpgroup 0 writes) and lo (warpgroup 1 writes)
-  {
-    const float* src = qbar + ((size_t)pq * dm.Cq + (i < dm.Cq ? i : 0)) * D;
-#pragma unroll
-    for (int ck = 0; ck < D / 8; ++ck) {
-      const float4 f0 = i < dm.Cq ? ld4(src + ck * 8) : make_float4(0.f, 0.f, 0.f, 0.f);
-      const float4 f1 = i < dm.Cq ? ld4(src + ck * 8 + 4) : make_float4(0.f, 0.f, 0.f, 0.f);
-      const float x[8] = {f0.x * dm.sigma, f0.y * dm.sigma, f0.z * dm.sigma, f0.w * dm.sigma,
-                          f1.x * dm.sigma, f1.y * dm.sigma, f1.z * dm.sigma, f1.w * dm.sigma};
-      uint32_t w[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        __nv_bfloat162 hh = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]);
-        __nv_bfloat162 ll = __floats2bfloat162_rn(x[2 * e] - __low2float(hh), x[2 * e + 1] - __high2float(hh));
-        w[e] = wg == 0 ? *reinterpret_cast<uint32_t*>(&hh) : *reinterpret_cast<uint32_t*>(&ll);
-      }
-      *reinterpret_cast<uint4*>(sm + (wg == 0 ? oQhi : oQlo) + (ck >> 3) * TI * 128 + tc::sw128_off(row, ck & 7)) = make_uint4(w[0], w[1], w[2], w[3]);
-    }
-  }
-  tc::fence_async_smem();
+  if (tid == 0) { tc::mbar_init(&bar_kv, 1); tc::mbar_init(&bar_q, 1); tc::mbar_init(&bar1, 1); tc::mbar_init(&bar2, 1); tc::mbar_init_fence(); }
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
+  // sigma * qbar tile as bf16 hi and lo operands, split once per layer and loaded here by TMA
+  if (tid == 0) {
+    tc::mbar_expect_tx(&bar_q, 2 * kTile);
+    const int r = pq * dm.Cq + i0;
+    tc::tma_load_2d(sm + oQhi, &tm_qhi, 0, r, &bar_q); tc::tma_load_2d(sm + oQhi + TI * 128, &tm_qhi, 64, r, &bar_q);
+    tc::tma_load_2d(sm + oQlo, &tm_qlo, 0, r, &bar_q); tc::tma_load_2d(sm + oQlo + TI * 128, &tm_qlo, 64, r, &bar_q);
+  }
   const uint32_t tbase = tbase_s, tlane = tbase + ((uint32_t)((warp & 3) * 32) << 16);
   const uint32_t aQhi = tc::smem_u32(sm + oQhi), aQlo = tc::smem_u32(sm + oQlo), aK = tc::smem_u32(sm + oK),
                  aV = tc::smem_u32(sm + oV), aWhi = tc::smem_u32(sm + oWhi), aWlo = tc::smem_u32(sm + oWlo);
   uint32_t ph_kv = 0, ph1 = 0, ph2 = 0;
-  bool ok = true;
+  bool ok = true, q_ready = false;
   float acc[D];
 #pragma unroll
   for (int d = 0; d < D; ++d) acc[d] = 0.f;
@@ -112,6 +117,7 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
       __syncthreads();
       const int ng = (nk + 15) >> 4;
       if (tid == 0) {
+        if (!q_ready) { if (!tc::mbar_wait(&bar_q, 0)) ok = false; q_ready = true; }
         if (!tc::mbar_wait(&bar_kv, ph_kv)) ok = false;
         tc::fence_after_sync();
         const uint32_t idesc = tc::idesc_bf16(TI, 16 * ng, 0, 0);
@@ -253,7 +259,16 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
 bool summarize_tc_supported(const Dims& d, int dtype) { return dtype == MUSE_BF16 && d.D == st::D; }
 
 int summarize_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const float* qbar, const SummPtrs& sp,
-                 int* status, cudaStream_t stream) {
+                 void* qsplit, int* status, cudaStream_t stream) {
+  // qsplit: 2 * B*Hq*Cq*D bf16 of scratch for the split centroids
+  bf16* qhi = (bf16*)qsplit;
+  bf16* qlo = qhi + (size_t)d.B * d.Hq * d.Cq * st::D;
+  int rcq = split_qbar(d, qbar, qhi, qlo, stream);
+  if (rcq != MUSE_OK) return rcq;
+  CUtensorMap tqh, tql;
+  rcq = make_tmap_bf16_rows(&tqh, qhi, (uint64_t)d.B * d.Hq * d.Cq, st::D, st::TI);
+  if (rcq == MUSE_OK) rcq = make_tmap_bf16_rows(&tql, qlo, (uint64_t)d.B * d.Hq * d.Cq, st::D, st::TI);
+  if (rcq != MUSE_OK) return rcq;
   CUtensorMap tK, tV;
   int rc = make_tmap_bf16_rows(&tK, Kp, (uint64_t)d.B * d.Hkv * d.N, st::D, 16);       // boxes of 16 keys
   if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tV, Vp, (uint64_t)d.B * d.Hkv * d.N, st::D, 16);
@@ -268,7 +283,7 @@ int summarize_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* o
   if (rc != MUSE_OK) return rc;
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, st::total));
   prof_mark("k_summarize_tc", stream);
-  k_summarize_tc<<<dim3(d.Ck, cdiv(d.Cq, st::TI), d.B * d.Hq), st::THREADS, st::total, stream>>>(d, tK, tV, okhi, oklo, onu, off_k, qbar, sp, status);
+  k_summarize_tc<<<dim3(d.Ck, cdiv(d.Cq, st::TI), d.B * d.Hq), st::THREADS, st::total, stream>>>(d, tK, tV, okhi, oklo, onu, tqh, tql, off_k, sp, status);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }
