@@ -65,6 +65,55 @@ k_sort_scan(int32_t* __restrict__ cnt, int nkeys, int nchunks, int32_t* __restri
   if (tid == 1023) o[nkeys] = run;     // the last thread ends on the grand total
 }
 
+// Same scan for the large [key][chunk] arrays of the bucket sorts: a problem's array is cut into
+// kScanParts contiguous parts, one CTA each.  The CTA first adds up everything in front of its part
+// (coalesced), then scans its part; the result goes to a second array because other CTAs still
+// read the counts.
+constexpr int kScanParts = 8;
+
+__global__ void __launch_bounds__(1024)
+k_sort_scan_parts(const int32_t* __restrict__ cnt, int32_t* __restrict__ pre, int nkeys, int nchunks, int32_t* __restrict__ off) {
+  __shared__ int32_t part[1024];
+  __shared__ int32_t base_s;
+  const int prob = blockIdx.x, g = blockIdx.y, tid = threadIdx.x;
+  const int L = nkeys * nchunks;
+  const int32_t* c = cnt + (size_t)prob * L;
+  int32_t* out = pre + (size_t)prob * L;
+  int32_t* o = off + (size_t)prob * (nkeys + 1);
+  const int plen = cdiv(L, kScanParts), p0 = min(L, g * plen), p1 = min(L, p0 + plen);
+  int s0 = 0;
+  for (int e = tid; e < p0; e += 1024) s0 += c[e];
+  part[tid] = s0;
+  __syncthreads();
+  for (int ofs = 512; ofs > 0; ofs >>= 1) {
+    if (tid < ofs) part[tid] += part[tid + ofs];
+    __syncthreads();
+  }
+  if (tid == 0) base_s = part[0];
+  __syncthreads();
+  const int base = base_s;
+  const int per = cdiv(p1 - p0, 1024);
+  const int e0 = min(p1, p0 + tid * per), e1 = min(p1, e0 + per);
+  int s = 0;
+  for (int e = e0; e < e1; ++e) s += c[e];
+  part[tid] = s;
+  __syncthreads();
+  for (int ofs = 1; ofs < 1024; ofs <<= 1) {       // Hillis-Steele inclusive scan
+    int v = tid >= ofs ? part[tid - ofs] : 0;
+    __syncthreads();
+    part[tid] += v;
+    __syncthreads();
+  }
+  int run = base + part[tid] - s;
+  for (int e = e0; e < e1; ++e) {
+    int v = c[e];
+    out[e] = run;
+    if (e % nchunks == 0) o[e / nchunks] = run;
+    run += v;
+  }
+  if (g == kScanParts - 1 && tid == 1023) o[nkeys] = run;     // the last thread of the last part ends on the grand total
+}
+
 int launch_scan(int32_t* cnt, int problems, int nkeys, int nchunks, int32_t* off, cudaStream_t st) {
   prof_mark("k_sort_scan", st);
   k_sort_scan<<<problems, 1024, 0, st>>>(cnt, nkeys, nchunks, off);
@@ -105,7 +154,8 @@ k_sort_scatter(const int32_t* __restrict__ assign, int N, int C, int S, int Bs, 
   }
 }
 
-size_t sort_ws_elems(int N, int nkeys) { return (size_t)nkeys * cdiv(N, kSortChunk); }
+// counts [key][chunk] and their exclusive scan
+size_t sort_ws_elems(int N, int nkeys) { return 2 * (size_t)nkeys * cdiv(N, kSortChunk); }
 
 int bucket_sort(int, const int32_t* assign, int problems, int N, int C, int S, int Bs, int kind,
                 int32_t* off, int32_t* perm, int32_t* scratch, cudaStream_t st) {
@@ -118,9 +168,12 @@ int bucket_sort(int, const int32_t* assign, int problems, int N, int C, int S, i
   prof_mark("k_sort_hist", st);
   k_sort_hist<<<dim3(nchunks, problems), kSortThreads, smem, st>>>(assign, N, C, S, Bs, kind, nkeys, nchunks, scratch);
   MUSE_LAUNCH_OK();
-  if (launch_scan(scratch, problems, nkeys, nchunks, off, st) != MUSE_OK) return MUSE_ERR_CUDA;
+  int32_t* pre = scratch + (size_t)problems * nkeys * nchunks;
+  prof_mark("k_sort_scan", st);
+  k_sort_scan_parts<<<dim3(problems, kScanParts), 1024, 0, st>>>(scratch, pre, nkeys, nchunks, off);
+  MUSE_LAUNCH_OK();
   prof_mark("k_sort_scatter", st);
-  k_sort_scatter<<<dim3(nchunks, problems), kSortThreads, smem, st>>>(assign, N, C, S, Bs, kind, nkeys, nchunks, scratch, perm);
+  k_sort_scatter<<<dim3(nchunks, problems), kSortThreads, smem, st>>>(assign, N, C, S, Bs, kind, nkeys, nchunks, pre, perm);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }
