@@ -5,6 +5,7 @@
 //   P  = softmax piece, one thread per row straight out of TMEM, written back as bf16 to smem
 //   PV              tcgen05.mma, A = P tile (K-major), B = V tile (MN-major), read from TMEM
 //                   and folded into the fp32 output registers with the online-softmax rescale.
+#include <cuda.h>
 #include "common.cuh"
 #include "tc05.cuh"
 
@@ -168,25 +169,34 @@ __device__ __forceinline__ void tc_teardown(TcCtx& c, int tid, int* status) {
 // ---- local (block-diagonal) attention ------------------------------------------------------------
 // 256 threads: thread (row, warpgroup w) owns key columns [32 w, 32 w + 32) of every 64-key tile and
 // output dims [D/2 w, D/2 w + D/2) of its row; the two halves of a row share the running maximum
-// through shared memory.  The next K / V tile is loaded into registers while the current one is on
-// the tensor core.
+// through shared memory.  Software pipeline over the key tiles t (K and V tiles arrive by TMA):
+//   S(t+1) = Q K_{t+1}^T is issued as soon as S(t) has landed (two S buffers in TMEM, two K tiles in
+//   shared memory), so it runs while the threads do the softmax of tile t; O(t) = P(t) V_t is
+//   collected at the start of iteration t + 1, which frees P and V for tile t + 1.
 constexpr int kLfThreads = 256;
+
+template <int D> struct LfSmem {
+  static constexpr int q = 0, k = q + kTcM * D * 2, v = k + 2 * kTcN * D * 2, p = v + kTcN * D * 2, total = p + kTcM * kTcN * 2 + 1024;
+};
 
 template <int D>
 __global__ void __launch_bounds__(kLfThreads, 2)
-k_local_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ K, const bf16* __restrict__ V,
-               float* __restrict__ o_loc, float* __restrict__ lse_loc, int* __restrict__ status) {
+k_local_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+               const bf16* __restrict__ Q, float* __restrict__ o_loc, float* __restrict__ lse_loc, int* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char sm_raw[];
-  __shared__ uint64_t bar[2];
+  __shared__ uint64_t barS[2], barK[2], barV, barPV;
   __shared__ uint32_t tbase_s;
   __shared__ float mx_s[2][kTcM];
-  constexpr int NKV = kTcN * (D / 8) / kLfThreads;         // 16-byte chunks of a K (or V) tile per thread
-  constexpr int HD = D / 2;
+  constexpr int HD = D / 2, kKB = kTcN * D * 2;
+  constexpr uint32_t cO = 2 * kTcN;                        // TMEM: S0 | S1 | O
   const int tid = threadIdx.x, warp = tid >> 5, row = tid & 127, wg = tid >> 7;
   unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
-  unsigned char *Qs = sm, *Ks = Qs + FwdTcSmem<D>::q_bytes, *Vs = Ks + FwdTcSmem<D>::k_bytes, *Ps = Vs + FwdTcSmem<D>::v_bytes;
-  if (warp == 0) tc::tmem_alloc(&tbase_s, D == 128 ? 256 : 128);
-  if (tid == 0) { tc::mbar_init(&bar[0], 1); tc::mbar_init(&bar[1], 1); tc::mbar_init_fence(); }
+  unsigned char *Qs = sm + LfSmem<D>::q, *Ks = sm + LfSmem<D>::k, *Vs = sm + LfSmem<D>::v, *Ps = sm + LfSmem<D>::p;
+  if (warp == 0) tc::tmem_alloc(&tbase_s, 256);
+  if (tid == 0) {
+    tc::mbar_init(&barS[0], 1); tc::mbar_init(&barS[1], 1); tc::mbar_init(&barK[0], 1); tc::mbar_init(&barK[1], 1);
+    tc::mbar_init(&barV, 1); tc::mbar_init(&barPV, 1); tc::mbar_init_fence();
+  }
   const int tpb = cdiv(dm.Bs, kTcM);
   // heaviest tiles (latest in a block) first
   const int lin = blockIdx.x, qt = tpb - 1 - lin / dm.S, blk = lin % dm.S, pq = blockIdx.y;
@@ -194,66 +204,76 @@ k_local_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ K, 
   const int bstart = blk * dm.Bs, bend = bstart + dm.Bs;
   const int q0 = bstart + qt * kTcM, nq = min(kTcM, bend - q0);
   const bf16* Qb = Q + (size_t)pq * dm.N * D;
-  const bf16* Kb = K + (size_t)pk * dm.N * D;
-  const bf16* Vb = V + (size_t)pk * dm.N * D;
+  const int k_lo = bstart, k_hi = q0 + nq;                  // causal: keys up to the tile's last row
+  const int T = (k_hi - k_lo + kTcN - 1) / kTcN;
+  const int krow0 = pk * dm.N + k_lo;                       // row of the first key in the [B*Hkv*N][D] tensors
   for (int e = tid; e < kTcM * (D / 8); e += kLfThreads) {
     const int r = e / (D / 8), ck = e % (D / 8);
     uint4 v = make_uint4(0u, 0u, 0u, 0u);
     if (r < nq) v = reinterpret_cast<const uint4*>(Qb + (size_t)(q0 + r) * D)[ck];
     *reinterpret_cast<uint4*>(Qs + (ck >> 3) * kTcM * 128 + tc::sw128_off(r, ck & 7)) = v;
   }
-  const int k_lo = bstart, k_hi = q0 + nq;                  // causal: keys up to the tile's last row
-  uint4 kreg[NKV], vreg[NKV];
-  auto load_kv = [&](int c0) {
-    const int nk = min(kTcN, k_hi - c0);
-#pragma unroll
-    for (int k = 0; k < NKV; ++k) {
-      const int e = tid + kLfThreads * k, r = e / (D / 8), ck = e % (D / 8);
-      kreg[k] = r < nk ? __ldg(reinterpret_cast<const uint4*>(Kb + (size_t)(c0 + r) * D) + ck) : make_uint4(0u, 0u, 0u, 0u);
-      vreg[k] = r < nk ? __ldg(reinterpret_cast<const uint4*>(Vb + (size_t)(c0 + r) * D) + ck) : make_uint4(0u, 0u, 0u, 0u);
-    }
-  };
-  load_kv(k_lo);
+  tc::fence_async_smem();
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
   const uint32_t tbase = tbase_s, tl = tbase + ((uint32_t)((warp & 3) * 32) << 16);
   const uint32_t qa = tc::smem_u32(Qs), ka = tc::smem_u32(Ks), va = tc::smem_u32(Vs), pa = tc::smem_u32(Ps);
+  bool ok = true;
+  // thread 0 only: tile loads and MMA issue.  Rows past the block's visible keys are loaded too (they are masked).
+  auto load_k = [&](int t) {
+    tc::mbar_expect_tx(&barK[t & 1], kKB);
+    for (int g = 0; g < D / 64; ++g) tc::tma_load_2d(Ks + (t & 1) * kKB + g * kTcN * 128, &tm_k, 64 * g, krow0 + t * kTcN, &barK[t & 1]);
+  };
+  auto load_v = [&](int t) {
+    tc::mbar_expect_tx(&barV, kKB);
+    for (int g = 0; g < D / 64; ++g) tc::tma_load_2d(Vs + g * kTcN * 128, &tm_v, 64 * g, krow0 + t * kTcN, &barV);
+  };
+  auto issue_s = [&](int t) {                               // S(t) = Q K_t^T into S buffer t & 1
+    if (!tc::mbar_wait(&barK[t & 1], (t >> 1) & 1)) ok = false;
+    tc::fence_after_sync();
+    const uint32_t idesc = tc::idesc_bf16(kTcM, kTcN, 0, 0);
+    const uint32_t kat = ka + (t & 1) * kKB;
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks)
+      tc::mma_bf16_ss(tbase + (t & 1) * kTcN, tc::smem_desc_sw128(qa + (ks / 4) * kTcM * 128 + (ks % 4) * 32, 16, 1024),
+                      tc::smem_desc_sw128(kat + (ks / 4) * kTcN * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
+    tc::mma_commit(&barS[t & 1]);
+  };
+  if (tid == 0) {
+    load_k(0);
+    if (T > 1) load_k(1);
+    issue_s(0);
+  }
   const float scale2 = dm.sigma * 1.4426950408889634f;
   const int my_limit = q0 + row;                            // last visible key of this row
   float o[HD], m2 = -INFINITY, l = 0.f;                     // l: this warpgroup's share of the row sum
 #pragma unroll
   for (int i = 0; i < HD; ++i) o[i] = 0.f;
-  uint32_t ph0 = 0, ph1 = 0;
-  bool ok = true;
-  for (int c0 = k_lo; c0 < k_hi && ok; c0 += kTcN) {
-    const int nk = min(kTcN, k_hi - c0);
-#pragma unroll
-    for (int k = 0; k < NKV; ++k) {
-      const int e = tid + kLfThreads * k, r = e / (D / 8), ck = e % (D / 8);
-      const uint32_t off = (ck >> 3) * kTcN * 128 + tc::sw128_off(r, ck & 7);
-      *reinterpret_cast<uint4*>(Ks + off) = kreg[k];
-      *reinterpret_cast<uint4*>(Vs + off) = vreg[k];
-    }
-    tc::fence_async_smem();
-    tc::fence_before_sync();
-    __syncthreads();
-    if (tid == 0) {
-      tc::fence_after_sync();
-      const uint32_t idesc = tc::idesc_bf16(kTcM, kTcN, 0, 0);
-#pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks)
-        tc::mma_bf16_ss(tbase, tc::smem_desc_sw128(qa + (ks / 4) * kTcM * 128 + (ks % 4) * 32, 16, 1024),
-                        tc::smem_desc_sw128(ka + (ks / 4) * kTcN * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
-      tc::mma_commit(&bar[0]);
-    }
-    __syncwarp();
-    if (c0 + kTcN < k_hi) load_kv(c0 + kTcN);               // next tile: loads fly during the products and the softmax
-    if (!tc::mbar_wait(&bar[0], ph0)) { ok = false; break; }
-    ph0 ^= 1;
+  auto collect = [&](int t) {                               // O(t) has landed: add this thread's half row
+    if (!tc::mbar_wait(&barPV, t & 1)) ok = false;
     tc::fence_after_sync();
+#pragma unroll
+    for (int d0 = 0; d0 < HD; d0 += 32) {
+      float v[32];
+      tc::tmem_ld32(tl + cO + wg * HD + d0, v);
+#pragma unroll
+      for (int i = 0; i < 32; ++i) o[d0 + i] += v[i];
+    }
+  };
+  for (int t = 0; t < T && ok; ++t) {
+    const int c0 = k_lo + t * kTcN, nk = min(kTcN, k_hi - c0);
+    if (!tc::mbar_wait(&barS[t & 1], (t >> 1) & 1)) { ok = false; break; }
+    tc::fence_after_sync();
+    if (tid == 0 && t + 1 < T) issue_s(t + 1);              // runs during this tile's softmax
+    __syncwarp();
+    if (t > 0) collect(t - 1);                              // frees P and V (thread 0 has seen the products complete)
+    if (tid == 0) {
+      load_v(t);
+      if (t + 2 < T) load_k(t + 2);                         // over K_t, which S(t) has consumed
+    }
     float s[32];
-    tc::tmem_ld32(tl + 32 * wg, s);
+    tc::tmem_ld32(tl + (t & 1) * kTcN + 32 * wg, s);
     const int vis = min(nk, my_limit - c0 + 1) - 32 * wg;  // visible columns among this thread's 32
     float mx = -INFINITY;
 #pragma unroll
@@ -264,47 +284,39 @@ k_local_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ K, 
     const float base = mn == -INFINITY ? 0.f : mn;
     const float resc = tc::fast_exp2(m2 - base);
     float rs = 0.f;
-    uint32_t pk[16];
 #pragma unroll
-    for (int i = 0; i < 32; i += 2) {
-      __nv_bfloat162 b = __floats2bfloat162_rn(tc::fast_exp2(s[i] - base), tc::fast_exp2(s[i + 1] - base));
-      rs += __low2float(b) + __high2float(b);               // the rounded values, as the P V product sees them
-      pk[i / 2] = *reinterpret_cast<uint32_t*>(&b);
+    for (int ch = 0; ch < 4; ++ch) {
+      uint32_t pk[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        __nv_bfloat162 b = __floats2bfloat162_rn(tc::fast_exp2(s[8 * ch + 2 * e] - base), tc::fast_exp2(s[8 * ch + 2 * e + 1] - base));
+        rs += __low2float(b) + __high2float(b);             // the rounded values, as the P V product sees them
+        pk[e] = *reinterpret_cast<uint32_t*>(&b);
+      }
+      *reinterpret_cast<uint4*>(Ps + tc::sw128_off(row, 4 * wg + ch)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
     }
     l = l * resc + rs;
     m2 = mn;
-#pragma unroll
-    for (int ch = 0; ch < 4; ++ch)
-      *reinterpret_cast<uint4*>(Ps + tc::sw128_off(row, 4 * wg + ch)) = make_uint4(pk[ch * 4], pk[ch * 4 + 1], pk[ch * 4 + 2], pk[ch * 4 + 3]);
-    tc::fence_async_smem();
-    tc::fence_before_sync();
-    __syncthreads();
-    if (tid == 0) {
-      tc::fence_after_sync();
-      const uint32_t idesc = tc::idesc_bf16(kTcM, D, 0, 1);
-#pragma unroll
-      for (int ks = 0; ks < kTcN / 16; ++ks)
-        tc::mma_bf16_ss(tbase + kTcN, tc::smem_desc_sw128(pa + ks * 32, 16, 1024),
-                        tc::smem_desc_sw128(va + ks * 16 * 128, kTcN * 128, 1024), idesc, ks > 0);
-      tc::mma_commit(&bar[1]);
-    }
-    __syncwarp();
     if (resc != 1.f) {
 #pragma unroll
       for (int i = 0; i < HD; ++i) o[i] *= resc;
     }
-    if (!tc::mbar_wait(&bar[1], ph1)) { ok = false; break; }
-    ph1 ^= 1;
-    tc::fence_after_sync();
-#pragma unroll
-    for (int d0 = 0; d0 < HD; d0 += 32) {
-      float v[32];
-      tc::tmem_ld32(tl + kTcN + wg * HD + d0, v);
-#pragma unroll
-      for (int i = 0; i < 32; ++i) o[d0 + i] += v[i];
-    }
+    tc::fence_async_smem();
     tc::fence_before_sync();
+    __syncthreads();
+    if (tid == 0) {
+      if (!tc::mbar_wait(&barV, t & 1)) ok = false;
+      tc::fence_after_sync();
+      const uint32_t idesc = tc::idesc_bf16(kTcM, D, 0, 1);
+#pragma unroll
+      for (int ks = 0; ks < kTcN / 16; ++ks)
+        tc::mma_bf16_ss(tbase + cO, tc::smem_desc_sw128(pa + ks * 32, 16, 1024),
+                        tc::smem_desc_sw128(va + ks * 16 * 128, kTcN * 128, 1024), idesc, ks > 0);
+      tc::mma_commit(&barPV);
+    }
+    __syncwarp();
   }
+  if (ok && T > 0) collect(T - 1);
   // the two halves of the row sum meet
   __syncthreads();
   mx_s[wg][row] = l;
@@ -320,7 +332,7 @@ k_local_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ K, 
   }
   tc::fence_before_sync();
   __syncthreads();
-  if (warp == 0) tc::tmem_dealloc(tbase, D == 128 ? 256 : 128);
+  if (warp == 0) tc::tmem_dealloc(tbase, 256);
   if (!ok && tid == 0) atomicExch(status, 1);
 }
 
@@ -669,17 +681,23 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   if (!ok_ && tid == 0) atomicExch(status, 1);
 }
 
+int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
+
 int local_fwd_tc(const Dims& d, const void* Q, const void* K, const void* V, float* o_loc, float* lse_loc, int* status,
                  cudaStream_t st) {
   const int pq = d.B * d.Hq;
+  CUtensorMap tk, tv;
+  int rc = make_tmap_bf16_rows(&tk, K, (uint64_t)d.B * d.Hkv * d.N, (uint32_t)d.D, kTcN);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tv, V, (uint64_t)d.B * d.Hkv * d.N, (uint32_t)d.D, kTcN);
+  if (rc != MUSE_OK) return rc;
   dim3 grid(d.S * cdiv(d.Bs, kTcM), pq);
   prof_mark("k_local_fwd_tc", st);
   if (d.D == 128) {
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_local_fwd_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdTcSmem<128>::total));
-    k_local_fwd_tc<128><<<grid, kLfThreads, FwdTcSmem<128>::total, st>>>(d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, o_loc, lse_loc, status);
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_local_fwd_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, LfSmem<128>::total));
+    k_local_fwd_tc<128><<<grid, kLfThreads, LfSmem<128>::total, st>>>(d, tk, tv, (const bf16*)Q, o_loc, lse_loc, status);
   } else {
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_local_fwd_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdTcSmem<64>::total));
-    k_local_fwd_tc<64><<<grid, kLfThreads, FwdTcSmem<64>::total, st>>>(d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, o_loc, lse_loc, status);
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_local_fwd_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, LfSmem<64>::total));
+    k_local_fwd_tc<64><<<grid, kLfThreads, LfSmem<64>::total, st>>>(d, tk, tv, (const bf16*)Q, o_loc, lse_loc, status);
   }
   MUSE_LAUNCH_OK();
   return MUSE_OK;
