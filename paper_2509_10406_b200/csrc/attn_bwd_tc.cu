@@ -8,6 +8,7 @@
 //   keys-on-M (dK, dV):  S^T = K Q^T, dP^T = V dO^T -> P^T, G^T -> dV += P^T dO, dK += G^T Q
 // Operand tiles are 128-byte-swizzled in shared memory; a [rows][D] tile serves both as a
 // K-major operand (contraction over D) and as an MN-major operand (contraction over rows).
+#include <cuda.h>
 #include "common.cuh"
 #include "tc05.cuh"
 
@@ -16,6 +17,7 @@
 namespace muse {
 
 typedef __nv_bfloat16 bf16;
+int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
 constexpr int kBM = 128, kBN = 64;
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -427,56 +429,171 @@ __device__ __forceinline__ void dkdv_step_tc(BwdCtx& c, const float* __restrict_
 
 constexpr int kKeysThreads = 256;       // keys-on-M kernels: two warpgroups share the 64 query columns
 
+// Local (block-diagonal) dK, dV: one CTA = 128 keys of a block against the query tiles (64 rows) that see
+// them.  Software pipeline over the query tiles t, all operand tiles by TMA:
+//   MMA1(t+1) (S^T = K Q^T, dP^T = V dO^T into the second accumulator buffer) is issued as soon as
+//   MMA1(t) has landed, so it runs while the threads turn S^T(t), dP^T(t) into P^T, G^T;
+//   MMA2(t) (dV += P^T dO, dK += G^T Q) runs during the next iteration; Q / dO tiles sit in a ring of
+//   three, refilled as soon as the MMAs that read a slot have completed.
+template <int D> struct LdkSmem {
+  static constexpr int k = 0, v = k + kBM * D * 2, qd = v + kBM * D * 2, tile = 2 * kBN * D * 2,       // ring slot = Q tile | dO tile
+                       pt = qd + 3 * tile, gt = pt + kBM * kBN * 2, total = gt + kBM * kBN * 2 + 1024;
+  static constexpr uint32_t cDV = 256, cDK = 256 + D, cols = 512;   // S^T / dP^T buffers at 0 / 64 and 128 / 192
+};
+
+// Warps 0-7 do the arithmetic; lane 0 of a ninth warp issues every TMA load and MMA, so that issuing never
+// delays a warp that the others wait for at the barriers.
+constexpr int kLdkThreads = kKeysThreads + 32, kLdkIssuer = kKeysThreads;
+
 template <int D>
-__global__ void __launch_bounds__(kKeysThreads)
-k_local_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ K, const bf16* __restrict__ V,
-                    const bf16* __restrict__ dO, const float* __restrict__ LSE, const float* __restrict__ delta,
+__global__ void __launch_bounds__(kLdkThreads, 1)
+k_local_bwd_dkdv_tc(Dims dm, const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_do,
+                    const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
+                    const float* __restrict__ LSE, const float* __restrict__ delta,
                     float* __restrict__ dK_orig, float* __restrict__ dV_orig, int* __restrict__ status) {
-  typedef KeysSmem<D> SM;
+  typedef LdkSmem<D> SM;
   extern __shared__ __align__(1024) unsigned char sm_raw[];
-  __shared__ uint64_t bar[2];
+  __shared__ uint64_t barKV, barQ[3], bar1[2], bar2;
   __shared__ uint32_t tbase_s;
-  __shared__ __align__(16) float Ls[kBN], ds[kBN];
-  const int tid = threadIdx.x, row = tid & 127, wg = tid >> 7;
-  BwdCtx c;
-  bwd_setup(c, sm_raw, bar, &tbase_s, SM::cols, tid);
-  const int tpb = cdiv(dm.Bs, kBM);
+  __shared__ __align__(16) float Ls[3][kBN], ds[3][kBN];
+  const int tid = threadIdx.x, warp = tid >> 5, row = tid & 127, wg = tid >> 7;
+  unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
+  if (warp == 0) tc::tmem_alloc(&tbase_s, SM::cols);
+  if (tid == 0) {
+    tc::mbar_init(&barKV, 1); tc::mbar_init(&bar2, 1);
+    for (int k = 0; k < 3; ++k) tc::mbar_init(&barQ[k], 1);
+    tc::mbar_init(&bar1[0], 1); tc::mbar_init(&bar1[1], 1);
+    tc::mbar_init_fence();
+  }
   const int lin = blockIdx.x, kt = lin / dm.S, blk = lin % dm.S, pq = blockIdx.y;   // early key tiles (most work) first
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int bstart = blk * dm.Bs, bend = bstart + dm.Bs;
   const int k0 = bstart + kt * kBM, nk = min(kBM, bend - k0);
-  const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
-  const bf16* Kb = K + (size_t)pk * dm.N * D; const bf16* Vb = V + (size_t)pk * dm.N * D;
-  fill_tile<D, kBM, kKeysThreads>(c.sm + SM::k, nk, [&](int r) { return Kb + (size_t)(k0 + r) * D; }, tid);
-  fill_tile<D, kBM, kKeysThreads>(c.sm + SM::v, nk, [&](int r) { return Vb + (size_t)(k0 + r) * D; }, tid);
-  bool started = false;
+  const int T = (bend - k0 + kBN - 1) / kBN;                // query tiles that see these keys
   const int u = k0 + row;
-  TileRegs<D, kBN, kKeysThreads> qreg, oreg;
-  float Lreg = 0.f, dreg = 0.f;
-  auto load_q = [&](int q0) {
-    const int nq = min(kBN, bend - q0);
-    tile_ldg<D, kBN, kKeysThreads>(qreg, nq, [&](int r) { return Qb + (size_t)(q0 + r) * D; }, tid);
-    tile_ldg<D, kBN, kKeysThreads>(oreg, nq, [&](int r) { return dOb + (size_t)(q0 + r) * D; }, tid);
-    if (tid < kBN) {
-      Lreg = tid < nq ? LSE[(size_t)pq * dm.N + q0 + tid] * kLog2e : 0.f;
-      dreg = tid < nq ? delta[(size_t)pq * dm.N + q0 + tid] : 0.f;
+  auto load_scalars = [&](int t) {                          // threads 0..63: L (log2 units) and delta of query tile t
+    if (tid < kBN && t < T) {
+      const int q = k0 + t * kBN + tid;
+      Ls[t % 3][tid] = q < bend ? LSE[(size_t)pq * dm.N + q] * kLog2e : 0.f;
+      ds[t % 3][tid] = q < bend ? delta[(size_t)pq * dm.N + q] : 0.f;
     }
   };
-  load_q(k0);
-  for (int q0 = k0; q0 < bend && c.ok; q0 += kBN) {
-    const int nq = min(kBN, bend - q0);
-    tile_sts<D, kBN, kKeysThreads>(qreg, c.sm + SM::q, tid);
-    tile_sts<D, kBN, kKeysThreads>(oreg, c.sm + SM::dO, tid);
-    if (tid < kBN) { Ls[tid] = Lreg; ds[tid] = dreg; }
-    dkdv_step_tc<D>(c, Ls, ds, [&](int col) { return col < nq && row < nk && u <= q0 + col; }, dm.sigma * kLog2e, started, tid,
-                    [&]() { if (q0 + kBN < bend) load_q(q0 + kBN); });
+  load_scalars(0); load_scalars(1); load_scalars(2);
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tbase = tbase_s, tl = tbase + ((uint32_t)((warp & 3) * 32) << 16);
+  const uint32_t ka = tc::smem_u32(sm + SM::k), va = tc::smem_u32(sm + SM::v), pa = tc::smem_u32(sm + SM::pt), ga = tc::smem_u32(sm + SM::gt);
+  bool ok = true;
+  // thread 0 only
+  auto load_qd = [&](int t) {
+    unsigned char* slot = sm + SM::qd + (t % 3) * SM::tile;
+    tc::mbar_expect_tx(&barQ[t % 3], SM::tile);
+    const int r = pq * dm.N + k0 + t * kBN;
+    for (int g = 0; g < D / 64; ++g) {
+      tc::tma_load_2d(slot + g * kBN * 128, &tm_q, 64 * g, r, &barQ[t % 3]);
+      tc::tma_load_2d(slot + kBN * D * 2 + g * kBN * 128, &tm_do, 64 * g, r, &barQ[t % 3]);
+    }
+  };
+  auto issue1 = [&](int t) {                                // S^T(t) = K Q_t^T, dP^T(t) = V dO_t^T into accumulator buffer t & 1
+    if (!tc::mbar_wait(&barQ[t % 3], (t / 3) & 1)) ok = false;
+    tc::fence_after_sync();
+    const uint32_t qa = tc::smem_u32(sm + SM::qd + (t % 3) * SM::tile), da = qa + kBN * D * 2;
+    const uint32_t idesc = tc::idesc_bf16(kBM, kBN, 0, 0), cb = tbase + (t & 1) * 2 * kBN;
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(cb, desc_k<kBM>(ka, ks), desc_k<kBN>(qa, ks), idesc, ks > 0);
+#pragma unroll
+    for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(cb + kBN, desc_k<kBM>(va, ks), desc_k<kBN>(da, ks), idesc, ks > 0);
+    tc::mma_commit(&bar1[t & 1]);
+  };
+  if (tid == kLdkIssuer) {
+    tc::mbar_expect_tx(&barKV, 2 * kBM * D * 2);
+    for (int g = 0; g < D / 64; ++g) {
+      tc::tma_load_2d(sm + SM::k + g * kBM * 128, &tm_k, 64 * g, pk * dm.N + k0, &barKV);
+      tc::tma_load_2d(sm + SM::v + g * kBM * 128, &tm_v, 64 * g, pk * dm.N + k0, &barKV);
+    }
+    load_qd(0);
+    if (T > 1) load_qd(1);
+    if (T > 2) load_qd(2);
+    if (!tc::mbar_wait(&barKV, 0)) ok = false;
+    issue1(0);
   }
-  if (c.ok) {                                   // warpgroup 0 writes dV, warpgroup 1 writes dK
+  const float scale2 = dm.sigma * kLog2e;
+  for (int t = 0; t < T && ok; ++t) {
+    const int q0 = k0 + t * kBN, nq = min(kBN, bend - q0);
+    if (!tc::mbar_wait(&bar1[t & 1], (t >> 1) & 1)) { ok = false; break; }
+    tc::fence_after_sync();
+    if (tid == kLdkIssuer && t + 1 < T) issue1(t + 1);       // runs while this tile's P^T, G^T are computed
+    __syncwarp();
+    float p[32], g[32];
+    if (warp < 8) {
+      float s[32], dp[32];
+      tc::tmem_ld32(tl + (t & 1) * 2 * kBN + 32 * wg, s);
+      tc::tmem_ld32(tl + (t & 1) * 2 * kBN + kBN + 32 * wg, dp);
+      const float* Lt = Ls[t % 3] + 32 * wg;
+      const float* dt = ds[t % 3] + 32 * wg;
+#pragma unroll
+      for (int k = 0; k < 8; ++k) {
+        const float4 a = *reinterpret_cast<const float4*>(Lt + 4 * k), b = *reinterpret_cast<const float4*>(dt + 4 * k);
+        const float Lc[4] = {a.x, a.y, a.z, a.w}, dc[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int col = 32 * wg + 4 * k + e;
+          const float ev = tc::fast_exp2(s[4 * k + e] * scale2 - Lc[e]);
+          const float pv = (col < nq && row < nk && u <= q0 + col) ? ev : 0.f;
+          p[4 * k + e] = pv;
+          g[4 * k + e] = pv * (dp[4 * k + e] - dc[e]);
+        }
+      }
+    }
+    if (t > 0) {                                            // MMA2(t - 1) has completed: P^T / G^T and its ring slot are free
+      if (!tc::mbar_wait(&bar2, (t - 1) & 1)) { ok = false; break; }
+      tc::fence_after_sync();
+      if (tid == kLdkIssuer && t + 2 < T) load_qd(t + 2);
+      load_scalars(t + 2);
+    }
+    if (warp < 8) {
+      store_row32(sm + SM::pt, row, wg, p);
+      store_row32(sm + SM::gt, row, wg, g);
+    }
+    tc::fence_async_smem();
+    tc::fence_before_sync();
+    __syncthreads();
+    if (tid == kLdkIssuer) {
+      tc::fence_after_sync();
+      const uint32_t qa = tc::smem_u32(sm + SM::qd + (t % 3) * SM::tile), da = qa + kBN * D * 2;
+      const uint32_t idesc = tc::idesc_bf16(kBM, D, 0, 1);
+#pragma unroll
+      for (int ks = 0; ks < kBN / 16; ++ks)
+        tc::mma_bf16_ss(tbase + SM::cDV, tc::smem_desc_sw128(pa + ks * 32, 16, 1024), desc_mn<kBN>(da, ks), idesc, t > 0 || ks > 0);
+#pragma unroll
+      for (int ks = 0; ks < kBN / 16; ++ks)
+        tc::mma_bf16_ss(tbase + SM::cDK, tc::smem_desc_sw128(ga + ks * 32, 16, 1024), desc_mn<kBN>(qa, ks), idesc, t > 0 || ks > 0);
+      tc::mma_commit(&bar2);
+    }
+    __syncwarp();
+  }
+  if (ok && T > 0) { if (!tc::mbar_wait(&bar2, (T - 1) & 1)) ok = false; }
+  tc::fence_after_sync();
+  if (warp < 8) {                                           // warpgroup 0 writes dV, warpgroup 1 writes dK (all their threads run the TMEM loads)
     const size_t at = ((size_t)pq * dm.N + k0 + row) * D;
-    if (wg == 0) read_acc_row<D>(c, 2 * kBN, 1.f, dV_orig + at, row < nk, tid);
-    else read_acc_row<D>(c, 2 * kBN + D, dm.sigma, dK_orig + at, row < nk, tid);
+    float* dst = (wg == 0 ? dV_orig : dK_orig) + at;
+    const float f = wg == 0 ? 1.f : dm.sigma;
+#pragma unroll
+    for (int d0 = 0; d0 < D; d0 += 32) {
+      float v[32];
+      tc::tmem_ld32(tl + (wg == 0 ? SM::cDV : SM::cDK) + d0, v);
+      if (ok && row < nk) {
+#pragma unroll
+        for (int i = 0; i < 32; i += 4)
+          *reinterpret_cast<float4*>(dst + d0 + i) = make_float4(v[i] * f, v[i + 1] * f, v[i + 2] * f, v[i + 3] * f);
+      }
+    }
   }
-  bwd_teardown(c, SM::cols, tid, status);
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tbase, SM::cols);
+  if (!ok && tid == 0) atomicExch(status, 2);
 }
 
 // One CTA per (key cluster j, plane, split, head): 128-key tiles of the run the plane sees, fed with
@@ -893,9 +1010,14 @@ int local_bwd_tc(const Dims& d, const void* Q, const void* K, const void* V, con
                  const float* delta, float* dQacc, float* dK_orig, float* dV_orig, int* status, cudaStream_t st) {
   const int pq = d.B * d.Hq;
   dim3 grid(d.S * cdiv(d.Bs, kBM), pq);
+  CUtensorMap tq, tdo, tk, tv;
+  int rc = make_tmap_bf16_rows(&tq, Q, (uint64_t)pq * d.N, (uint32_t)d.D, kBN);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tdo, dO, (uint64_t)pq * d.N, (uint32_t)d.D, kBN);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tk, K, (uint64_t)d.B * d.Hkv * d.N, (uint32_t)d.D, kBM);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tv, V, (uint64_t)d.B * d.Hkv * d.N, (uint32_t)d.D, kBM);
+  if (rc != MUSE_OK) return rc;
   prof_mark("k_local_bwd_dkdv_tc", st);
-  MUSE_TC_LAUNCH(k_local_bwd_dkdv_tc, KeysSmem, kKeysThreads, grid, d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, (const bf16*)dO, LSE,
-                 delta, dK_orig, dV_orig, status);
+  MUSE_TC_LAUNCH(k_local_bwd_dkdv_tc, LdkSmem, kLdkThreads, grid, d, tq, tdo, tk, tv, LSE, delta, dK_orig, dV_orig, status);
   prof_mark("k_local_bwd_dq_tc", st);
   MUSE_TC_LAUNCH(k_local_bwd_dq_tc, RowsSmem, kRowsThreads, grid, d, (const bf16*)Q, (const bf16*)K, (const bf16*)V, (const bf16*)dO, LSE,
                  delta, dQacc, status);
