@@ -20,7 +20,8 @@ namespace muse {
 typedef __nv_bfloat16 bf16;
 
 namespace sb {
-constexpr int D = 128, TI = 128, NU = 64, THREADS = 256;
+constexpr int D = 128, TI = 128, NU = 64;
+constexpr int THREADS = 288, ISSUER = 256;     // warps 0-7 do the arithmetic; lane 0 of a ninth warp issues every TMA load and MMA
 constexpr int kTile = TI * D * 2;              // 32 KB
 constexpr int kKeys = NU * D * 2;              // 16 KB
 // The low half of the centroid tile is only needed for the tilt logits, which do not depend on
@@ -48,6 +49,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
   const int j = blockIdx.x, pq = blockIdx.y;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int tid = threadIdx.x, warp = tid >> 5, wg = tid >> 7, L = tid & 127;
+  const bool cw = warp < 8;                               // compute warp (the ninth warp only issues)
   const int32_t* ok_ = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const int32_t* oq = off_q + (size_t)pq * (dm.S * dm.Cq + 1);
   const int kbeg = ok_[0];
@@ -77,7 +79,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
 #endif
   for (int c0 = kbeg; c0 < kvis && ok; c0 += NU) {        // 64 keys of the cluster at a time (usually one chunk)
     __syncthreads();
-    if (tid == 0) {
+    if (tid == ISSUER) {
       tc::mbar_expect_tx(&bar_kv, 2 * kKeys);
       const int row = (int)((size_t)pk * dm.N + c0);
       tc::tma_load_2d(sm + oK, &tm_K, 0, row, &bar_kv); tc::tma_load_2d(sm + oK + NU * 128, &tm_K, 64, row, &bar_kv);
@@ -90,7 +92,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
     bool started = false;                                 // dK^T / dV^T accumulate in TMEM over all (i tile, plane)
     for (int i0 = 0; i0 < dm.Cq && ok; i0 += TI) {
       const int i = i0 + L;
-      const bool in_range = i < dm.Cq;
+      const bool in_range = cw && i < dm.Cq;
       const int ic = in_range ? i : 0;
       auto issue_grad = [&](int pl, int buf) {            // thread 0: both gradient tiles of (plane, j, i0..i0+127)
         tc::mbar_expect_tx(&bar_g[buf], 2 * kTile);
@@ -102,7 +104,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
       };
       PCLK(7)
       __syncthreads();                                    // every MMA that read the centroid tiles has completed (bar2 waited)
-      if (tid == 0) {
+      if (tid == ISSUER) {
         // sigma * qbar tile as bf16 hi + lo operands (split once per layer), and the first gradient tiles
         tc::mbar_expect_tx(&bar_q, 2 * kTile);
         const int r = pq * dm.Cq + i0;
@@ -117,7 +119,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         if (in_range && oq[(size_t)blk * dm.Cq + i + 1] > oq[(size_t)blk * dm.Cq + i]) livemask |= 1u << pl;
       }
       // tilt logits l_iu = sigma qbar_i . k_u, the same for every plane: once per centroid tile
-      if (tid == 0) {
+      if (tid == ISSUER) {
         if (!tc::mbar_wait(&bar_q, ph_q)) ok = false;
         tc::fence_after_sync();
         const uint32_t idesc = tc::idesc_bf16(TI, NU, 0, 0);
@@ -138,7 +140,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
       tc::fence_after_sync();
       PCLK(0)
       float lg[32];
-      tc::tmem_ld32(tlane + cL + 32 * wg, lg);            // this thread's logits: row i, keys 32 wg .. 32 wg + 31
+      if (cw) tc::tmem_ld32(tlane + cL + 32 * wg, lg);            // this thread's logits: row i, keys 32 wg .. 32 wg + 31
       // per-plane scalars, loaded one plane ahead
       auto ent_of = [&](int pl) { return (((size_t)pq * dm.SB + pl) * dm.Cq + ic) * dm.Ck + j; };        // summaries: [plane][i][j]
       auto gent_of = [&](int pl) { return (((size_t)pq * dm.SB + pl) * dm.Ck + j) * dm.Cq + ic; };      // gradients: [plane][j][i]
@@ -155,14 +157,14 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
           tc::fence_after_sync();
         }
         PCLK(1)
-        if (tid == 0 && pl + 1 < dm.SB && ok) issue_grad(pl + 1, buf ^ 1);
+        if (tid == ISSUER && pl + 1 < dm.SB && ok) issue_grad(pl + 1, buf ^ 1);
         if (pl + 1 < dm.SB && ((livemask >> (pl + 1)) & 1u)) { mu_n = mu[ent_of(pl + 1)]; dS_n = dS[gent_of(pl + 1)]; }
         if (!tc::mbar_wait(&bar_g[buf], ph_g[buf])) ok = false;
         ph_g[buf] ^= 1;
         PCLK(2)
         const int oDka = buf ? oQlo : oDka0, oDnu = buf ? oDnu1 : oDnu0;
         // rows of query clusters whose segment is empty (or beyond Cq) were never written: clear them
-        if (!live) {
+        if (cw && !live) {
 #pragma unroll
           for (int c8 = 0; c8 < D / 16; ++c8) {
             const int ck = wg * (D / 16) + c8;
@@ -175,7 +177,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         tc::fence_before_sync();
         __syncthreads();
         const uint32_t aDka = tc::smem_u32(sm + oDka), aDnu = tc::smem_u32(sm + oDnu);
-        if (tid == 0) {
+        if (tid == ISSUER) {
           tc::fence_after_sync();
           const uint32_t idesc = tc::idesc_bf16(TI, NU, 0, 0);
 #pragma unroll
@@ -193,7 +195,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         ph1 ^= 1;
         tc::fence_after_sync();
         PCLK(3)
-        {
+        if (cw) {
           float x1[32], x2[32];
           tc::tmem_ld32(tlane + cX1 + 32 * wg, x1);
           tc::tmem_ld32(tlane + cX2 + 32 * wg, x2);
@@ -215,7 +217,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         tc::fence_async_smem();
         tc::fence_before_sync();
         __syncthreads();
-        if (tid == 0) {
+        if (tid == ISSUER) {
           tc::fence_after_sync();
           const uint32_t idesc = tc::idesc_bf16(D, NU, 1, 1);       // A [i][d] and B [i][u]: both contract over rows
 #pragma unroll
@@ -250,7 +252,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
     PCLK(5)
     // read-out once per key chunk: thread = d, warpgroup = half of the keys; add into the fp32 accumulators
     const int nkc = min(NU, kvis - c0);
-    {
+    if (cw) {
       float a[32], b[32];
       tc::tmem_ld32(tlane + cDK + 32 * wg, a);
       tc::tmem_ld32(tlane + cDV + 32 * wg, b);
