@@ -1,8 +1,8 @@
 // Accumulated tilted summaries on the tensor cores (bf16 mode, D = 128): Eq. 3-5 and the
 // exclusive causal accumulation of Algorithm 1 in one online-softmax walk over the buckets of a
 // key cluster.  One CTA = (key cluster j, 128 query clusters, head), 256 threads: thread
-// (row i, warpgroup w) keeps the running max / mass of centroid i and 128 fp32 accumulators —
-// the kappa half (w = 0) or the nu half (w = 1).
+// (row i, warpgroup w) keeps the running max / mass of centroid i and 128 fp32 accumulators:
+// dims [64 w, 64 w + 64) of kappa and of nu.
 //   L   = sigma qbar K^T        tcgen05, qbar as bf16 hi + lo, keys TMA-loaded 64 at a time
 //   w_u = exp(l_u - running max)  per thread, written as a bf16 hi + lo operand pair
 //   U   = W [K | V]             tcgen05 (keys contracted), folded into the accumulators with the
@@ -191,9 +191,9 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
       if (tid == 0 && ok) issue_after(c0 + nk);          // key / value tiles are free again
       PCLK(3)
 #pragma unroll
-      for (int d0 = 0; d0 < D; d0 += 32) {
+      for (int d0 = 0; d0 < D; d0 += 32) {              // acc[0..63]: kappa dims 64 wg.., acc[64..127]: nu dims 64 wg..
         float v[32];
-        tc::tmem_ld32(tlane + (wg == 0 ? cUk : cUv) + d0, v);
+        tc::tmem_ld32(tlane + (d0 < D / 2 ? cUk : cUv) + (D / 2) * wg + (d0 & (D / 2 - 1)), v);
 #pragma unroll
         for (int e = 0; e < 32; ++e) acc[d0 + e] = fmaf(acc[d0 + e], sc, v[e]);
       }
@@ -218,7 +218,7 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
     if (tid == 0) tc::tma_store_wait_read();                           // the previous plane's stores have read the tiles
     __syncthreads();
 #pragma unroll
-    for (int ck = 0; ck < D / 8; ++ck) {
+    for (int ck = 0; ck < D / 16; ++ck) {                // this warpgroup's half of the kappa row: hi and lo tiles
       uint32_t w[4], wl_[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
@@ -227,13 +227,19 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
         __nv_bfloat162 ll = __floats2bfloat162_rn(x0 - __low2float(hh), x1 - __high2float(hh));
         w[e] = *reinterpret_cast<uint32_t*>(&hh); wl_[e] = *reinterpret_cast<uint32_t*>(&ll);
       }
-      const uint32_t off = (ck >> 3) * TI * 128 + tc::sw128_off(row, ck & 7);
-      if (wg == 0) {
-        *reinterpret_cast<uint4*>(sm + oStage + off) = make_uint4(w[0], w[1], w[2], w[3]);
-        *reinterpret_cast<uint4*>(sm + oStage + kTile + off) = make_uint4(wl_[0], wl_[1], wl_[2], wl_[3]);
-      } else {
-        *reinterpret_cast<uint4*>(sm + oStage + 2 * kTile + off) = make_uint4(w[0], w[1], w[2], w[3]);
+      const uint32_t off = wg * TI * 128 + tc::sw128_off(row, ck);       // 64-column group wg of the tile
+      *reinterpret_cast<uint4*>(sm + oStage + off) = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(sm + oStage + kTile + off) = make_uint4(wl_[0], wl_[1], wl_[2], wl_[3]);
+    }
+#pragma unroll
+    for (int ck = 0; ck < D / 16; ++ck) {                // and its half of the nu row
+      uint32_t w[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        __nv_bfloat162 hh = __floats2bfloat162_rn(acc[D / 2 + ck * 8 + 2 * e] * inv, acc[D / 2 + ck * 8 + 2 * e + 1] * inv);
+        w[e] = *reinterpret_cast<uint32_t*>(&hh);
       }
+      *reinterpret_cast<uint4*>(sm + oStage + 2 * kTile + wg * TI * 128 + tc::sw128_off(row, ck)) = make_uint4(w[0], w[1], w[2], w[3]);
     }
     tc::fence_async_smem();
     __syncthreads();
