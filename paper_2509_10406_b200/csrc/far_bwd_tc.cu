@@ -22,7 +22,8 @@ int make_tmap_bf16_nd(void* out_map, const void* base, int rank, const uint64_t*
                       const uint32_t* box);
 
 namespace fb {
-constexpr int D = 128, TJ = 128, NR = 64, NP = 1, THREADS = 256;
+constexpr int D = 128, TJ = 128, NR = 64, NP = 1;
+constexpr int THREADS = 288, CW = 256, ISSUER = 256;   // warps 0-7 do the arithmetic; lane 0 of a ninth warp issues every TMA transfer and MMA
 constexpr int kTile = TJ * D * 2;                 // 32 KB operand tile [128][128] bf16
 constexpr int kRows = NR * D * 2;                 // 16 KB tile of 64 query rows
 constexpr int oHi = 0, oLo = oHi + kTile, oNu = oLo + kTile;
@@ -52,7 +53,9 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
              bf16* __restrict__ dnu, float* __restrict__ dS, int grad_by_key_cluster, int* __restrict__ status) {
   using namespace fb;
   extern __shared__ __align__(1024) unsigned char sm_raw[];
-  __shared__ uint64_t bar_full, bar1, bar2;
+  // bar_full: kappa tiles landed; bar_nu: nu tile landed; bar1: S / dPnu products done; bar2: dnu / dkappa
+  // products done; bar3: dq products done as well; bar_st: the previous tile's stores have read their staging
+  __shared__ uint64_t bar_full, bar_nu, bar1, bar2, bar3, bar_st;
   __shared__ uint32_t tbase_s;
   __shared__ int32_t rows[NP * NR];
   __shared__ __align__(16) float Ls[NP * NR], ds[NP * NR], qb[D], part[2][TJ], dsid[2][TJ];
@@ -70,13 +73,15 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   const int32_t* pm = perm_q + (size_t)pq * dm.N;
 
   if (warp == 0) tc::tmem_alloc(&tbase_s, 512);
-  if (tid == 0) { tc::mbar_init(&bar_full, 1); tc::mbar_init(&bar1, 1); tc::mbar_init(&bar2, 1); tc::mbar_init_fence(); }
+  if (tid == 0) { tc::mbar_init(&bar_full, 1); tc::mbar_init(&bar1, 1); tc::mbar_init(&bar2, 1); tc::mbar_init(&bar3, 1);
+                  tc::mbar_init(&bar_nu, 1); tc::mbar_init(&bar_st, 1); tc::mbar_init_fence(); }
   if (tid < D) qb[tid] = qbar[((size_t)pq * dm.Cq + i) * D + tid];
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
   const uint32_t tbase = tbase_s, tlane = tbase + ((uint32_t)((warp & 3) * 32) << 16);
-  uint32_t ph_full = 0, ph1 = 0, ph2 = 0;
+  uint32_t ph_full = 0, ph1 = 0, ph2 = 0, ph3 = 0, ph_st = 0;
+  const bool cw = warp < 8;                               // compute warp
   bool ok = true;
   const uint32_t aHi = tc::smem_u32(sm + oHi), aLo = tc::smem_u32(sm + oLo), aNu = tc::smem_u32(sm + oNu),
                  aPt = tc::smem_u32(sm + oPt), aGt = tc::smem_u32(sm + oGt);
@@ -114,17 +119,22 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     long long pc[6] = {0, 0, 0, 0, 0, 0};
 #endif
     float bnext = beta[ent0 + L];
-    auto issue_tile = [&](int jt_) {                        // thread 0: the three operand tiles of cluster tile jt_
-      tc::mbar_expect_tx(&bar_full, 3 * kTile);
+    auto issue_kappa = [&](int jt_) {                       // issuer: the two kappa tiles of cluster tile jt_
+      tc::mbar_expect_tx(&bar_full, 2 * kTile);
       const int row = (int)(ent0 + (size_t)jt_ * TJ);
       tc::tma_load_2d(sm + oHi, &tm_khi, 0, row, &bar_full); tc::tma_load_2d(sm + oHi + TJ * 128, &tm_khi, 64, row, &bar_full);
       tc::tma_load_2d(sm + oLo, &tm_klo, 0, row, &bar_full); tc::tma_load_2d(sm + oLo + TJ * 128, &tm_klo, 64, row, &bar_full);
-      tc::tma_load_2d(sm + oNu, &tm_nu, 0, row, &bar_full); tc::tma_load_2d(sm + oNu + TJ * 128, &tm_nu, 64, row, &bar_full);
+    };
+    auto issue_nu = [&](int jt_) {                          // issuer: its nu tile
+      tc::mbar_expect_tx(&bar_nu, kTile);
+      const int row = (int)(ent0 + (size_t)jt_ * TJ);
+      tc::tma_load_2d(sm + oNu, &tm_nu, 0, row, &bar_nu); tc::tma_load_2d(sm + oNu + TJ * 128, &tm_nu, 64, row, &bar_nu);
     };
     const bool later_sweep = s0 > p0;                       // gradients of earlier sweeps are already stored: add to them
-    if (tid == 0) {
+    if (tid == ISSUER) {
       if (later_sweep) tc::tma_store_wait_all();
-      issue_tile(0);
+      issue_kappa(0);
+      issue_nu(0);
     }
     if (later_sweep) __syncthreads();
     for (int jt = 0; jt < NJ && ok; ++jt) {
@@ -139,10 +149,10 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       const float mu1 = 1.f + mu[ent0 + j];                               // 1 + accumulated log-mass of cluster j
       for (int p = 0; p < np && ok; ++p) {
         const uint32_t aQ = tc::smem_u32(sm + oQ + p * kRows), aDO = tc::smem_u32(sm + oDO + p * kRows);
-        if (tid == 0) {
+        if (tid == ISSUER) {
           if (p == 0) {
             if (!tc::mbar_wait(&bar_full, ph_full)) ok = false;
-            tc::tma_store_wait_read();        // the previous tile's stores have read the P / G tiles, which are written again below
+            if (!tc::mbar_wait(&bar_nu, ph_full)) ok = false;
           }
           tc::fence_after_sync();
           const uint32_t idesc = tc::idesc_bf16(TJ, NR, 0, 0);
@@ -159,15 +169,20 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
             tc::mma_bf16_ss(tbase + cDP, tc::smem_desc_sw128(aNu + (ks / 4) * TJ * 128 + (ks % 4) * 32, 16, 1024),
                             tc::smem_desc_sw128(aDO + (ks / 4) * NR * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
           tc::mma_commit(&bar1);
+          if (p == 0) {
+            tc::tma_store_wait_read();        // the previous tile's stores have read the staging tiles, which the
+            tc::mbar_arrive(&bar_st);         // compute warps write again (P / G tiles first)
+          }
+          if (!tc::mbar_wait(&bar1, ph1)) ok = false;
+          if (p + 1 == np && jt + 1 < NJ && ok) issue_nu(jt + 1);     // the nu tile is only read by the products above
         }
-        __syncwarp();
-        if (!tc::mbar_wait(&bar1, ph1)) ok = false;
+        if (cw && !tc::mbar_wait(&bar1, ph1)) ok = false;
         ph1 ^= 1;
         tc::fence_after_sync();
 #ifdef MUSE_PHASE_CLOCKS
         if (p == 0) k1_ = clock64();
 #endif
-        {
+        if (cw) {
           float s[32], dp[32];
           tc::tmem_ld32(tlane + cS + 32 * wg, s);
           tc::tmem_ld32(tlane + cDP + 32 * wg, dp);
@@ -211,6 +226,10 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #ifdef MUSE_PHASE_CLOCKS
           if (p == 0 && tid == 0 && blockIdx.x == 5 && blockIdx.y == 3 && blockIdx.z == 0 && jt == 3) status[33] = (int)(clock64() - k1_);
 #endif
+          if (p == 0) {
+            if (!tc::mbar_wait(&bar_st, ph_st)) ok = false;
+            ph_st ^= 1;
+          }
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
             *reinterpret_cast<uint4*>(sm + oPt + tc::sw128_off(L, 4 * wg + ch)) = make_uint4(pw[4 * ch], pw[4 * ch + 1], pw[4 * ch + 2], pw[4 * ch + 3]);
@@ -223,7 +242,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
         tc::fence_async_smem();
         tc::fence_before_sync();
         __syncthreads();
-        if (tid == 0) {
+        if (tid == ISSUER) {
           tc::fence_after_sync();
           const uint32_t id_row = tc::idesc_bf16(TJ, D, 0, 1);      // A K-major (P / G), B = query rows, MN-major
           const uint32_t id_dq = tc::idesc_bf16(D, NR, 1, 1);       // A = kappa tile MN-major, B = G MN-major
@@ -235,6 +254,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
           for (int ks = 0; ks < NR / 16; ++ks)
             tc::mma_bf16_ss(tbase + cDKA, tc::smem_desc_sw128(aGt + ks * 32, 16, 1024),
                             tc::smem_desc_sw128(aQ + ks * 16 * 128, NR * 128, 1024), id_row, !(p == 0 && ks == 0));
+          tc::mma_commit(&bar2);              // the read-out of dnu / dkappa can start while the dq products still run
 #pragma unroll
           for (int ks = 0; ks < TJ / 16; ++ks)
             tc::mma_bf16_ss(tbase + cDQ + p * NR, tc::smem_desc_sw128(aHi + ks * 16 * 128, TJ * 128, 1024),
@@ -243,30 +263,38 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
           for (int ks = 0; ks < TJ / 16; ++ks)
             tc::mma_bf16_ss(tbase + cDQ + p * NR, tc::smem_desc_sw128(aLo + ks * 16 * 128, TJ * 128, 1024),
                             tc::smem_desc_sw128(aGt + ks * 16 * 128, TJ * 128, 1024), id_dq, 1);
-          tc::mma_commit(&bar2);
+          tc::mma_commit(&bar3);
+          // every MMA on the operand tiles has completed: the next cluster tile may overwrite them
+          if (!tc::mbar_wait(&bar3, ph3)) ok = false;
+          if (p + 1 == np && jt + 1 < NJ && ok) issue_kappa(jt + 1);
         }
-        __syncwarp();
-        if (!tc::mbar_wait(&bar2, ph2)) ok = false;
+        if (cw && !tc::mbar_wait(&bar2, ph2)) ok = false;
+        // a further pass writes the P / G tiles again: the dq products must have read them
+        if (cw && p + 1 < np && !tc::mbar_wait(&bar3, ph3)) ok = false;
         ph2 ^= 1;
+        ph3 ^= 1;
         tc::fence_after_sync();
       }
       ph_full ^= 1;
-      if (tid == 0 && jt + 1 < NJ && ok) issue_tile(jt + 1);    // every MMA on the operand tiles has completed
 #ifdef MUSE_PHASE_CLOCKS
       k3_ = clock64();
 #endif
       // ---- tile read-out: warpgroup 0 -> dnu, warpgroup 1 -> dkappa; both need sum_r g
-      part[wg][L] = gsum;
-      dsid[wg][L] = dsum;
-      __syncthreads();
-      const float gtot = part[0][L] + part[1][L];
+      float gtot = 0.f;
+      if (cw) {
+        part[wg][L] = gsum; dsid[wg][L] = dsum;
+        tc::named_bar_sync(1, CW);                          // the issuer is still waiting for the dq products
+        gtot = part[0][L] + part[1][L];
+      }
       // gradient entry: [plane][i][j] like the summaries, or [plane][j][i] so that the key-side
       // pass finds the 128 query clusters of one key cluster in one contiguous tile
       const size_t gent = grad_by_key_cluster ? (((size_t)pq * dm.SB + pl) * Ck + j) * dm.Cq + i : ent0 + j;
 #pragma unroll
-      for (int d0 = 0; d0 < D; d0 += 32) {
+      for (int d0 = 0; cw && d0 < D; d0 += 32) {
         float v[32];
         tc::tmem_ld32(tlane + (wg == 0 ? cDNU : cDKA) + d0, v);
+        // the second half of the dkappa staging is the G tile, which the dq products read
+        if (wg == 1 && d0 == 64 && !tc::mbar_wait(&bar3, ph3 ^ 1)) ok = false;
 #pragma unroll
         for (int ch = 0; ch < 4; ++ch) {
           const int d = d0 + 8 * ch;
@@ -299,7 +327,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       // [plane][j][i] layout (adjacent in the [plane][i][j] one)
       tc::fence_async_smem();
       __syncthreads();
-      if (tid == 0 && ok) {
+      if (tid == ISSUER && ok) {
         const int c1 = grad_by_key_cluster ? i : 0;
         const int c2 = grad_by_key_cluster ? (pq * dm.SB + pl) * Ck + jt * TJ : (int)(ent0 + (size_t)jt * TJ);
         tc::tma_store_3d(&tm_gnu, sm + oStN, 0, c1, c2); tc::tma_store_3d(&tm_gnu, sm + oStN + TJ * 128, 64, c1, c2);
@@ -318,9 +346,10 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       for (int k = 0; k < 6; ++k) status[24 + k] = (int)pc[k];
 #endif
     // ---- dq: warpgroup p reads pass p (thread = output dim), adds into the fp32 accumulator
-    for (int p = wg; p < np; p += 2) {
-#pragma unroll
-      for (int c0 = 0; c0 < NR; c0 += 32) {
+    if (cw && !tc::mbar_wait(&bar3, ph3 ^ 1)) ok = false;     // the last tile's dq products
+    tc::fence_after_sync();
+    for (int p = 0; cw && p < np; ++p) {
+      for (int c0 = 32 * wg; c0 < NR; c0 += 64) {
         float v[32];
         tc::tmem_ld32(tlane + cDQ + p * NR + c0, v);
         if (ok) {
@@ -336,7 +365,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   }
   tc::fence_before_sync();
   __syncthreads();
-  if (tid == 0) tc::tma_store_wait_all();
+  if (tid == ISSUER) tc::tma_store_wait_all();
   if (warp == 0) tc::tmem_dealloc(tbase, 512);
   if (!ok && tid == 0) atomicExch(status, 4);
 }
