@@ -86,16 +86,30 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   const uint32_t aHi = tc::smem_u32(sm + oHi), aLo = tc::smem_u32(sm + oLo), aNu = tc::smem_u32(sm + oNu),
                  aPt = tc::smem_u32(sm + oPt), aGt = tc::smem_u32(sm + oGt);
 
-  for (int s0 = p0; s0 < p1 && ok; s0 += NP * NR) {        // super-pass: up to 128 rows
+  auto issue_kappa = [&](int jt_) {                       // issuer: the two kappa tiles of cluster tile jt_
+    tc::mbar_expect_tx(&bar_full, 2 * kTile);
+    const int row = (int)(ent0 + (size_t)jt_ * TJ);
+    tc::tma_load_2d(sm + oHi, &tm_khi, 0, row, &bar_full); tc::tma_load_2d(sm + oHi + TJ * 128, &tm_khi, 64, row, &bar_full);
+    tc::tma_load_2d(sm + oLo, &tm_klo, 0, row, &bar_full); tc::tma_load_2d(sm + oLo + TJ * 128, &tm_klo, 64, row, &bar_full);
+  };
+  auto issue_nu = [&](int jt_) {                          // issuer: its nu tile
+    tc::mbar_expect_tx(&bar_nu, kTile);
+    const int row = (int)(ent0 + (size_t)jt_ * TJ);
+    tc::tma_load_2d(sm + oNu, &tm_nu, 0, row, &bar_nu); tc::tma_load_2d(sm + oNu + TJ * 128, &tm_nu, 64, row, &bar_nu);
+  };
+  for (int s0 = p0; s0 < p1 && ok; s0 += NP * NR) {        // sweep: up to 64 rows
     const int ns = min(NP * NR, p1 - s0), np = (ns + NR - 1) / NR;
     __syncthreads();
+    // the operand tiles are free (every product of the previous sweep has completed): the first cluster
+    // tile travels while the rows are gathered
+    if (tid == ISSUER) { issue_kappa(0); issue_nu(0); }
     if (tid < NP * NR) {
       const int t = tid < ns ? pm[s0 + tid] : -1;
       rows[tid] = t;
       Ls[tid] = t >= 0 ? LSE[(size_t)pq * dm.N + t] * kLog2e : 0.f;
       ds[tid] = t >= 0 ? delta[(size_t)pq * dm.N + t] : 0.f;
     }
-    for (int e = tid; e < NP * NR * MW; e += THREADS) smask[e] = 0u;
+    for (int e = tid; e < 2 * Ck; e += THREADS) smask[e] = 0u;
     __syncthreads();
     for (int e = tid; e < NP * NR * (D / 8); e += THREADS) {
       const int r = e >> 4, ck = e & 15, kb = ck >> 3, c = ck & 7, p = r / NR, rr = r % NR;
@@ -110,7 +124,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     for (int e = tid; e < ns * m; e += THREADS) {
       const int r = e / m, k = e % m;
       const int c = sel[((size_t)pq * dm.N + rows[r]) * m + k];
-      if (c >= 0 && c < Ck) atomicOr(&smask[(c >> 5) * (NP * NR) + r], 1u << (c & 31));     // [word][row]
+      if (c >= 0 && c < Ck) atomicOr(&smask[2 * c + (r >> 5)], 1u << (r & 31));     // [cluster][row bits]
     }
     tc::fence_async_smem();
     __syncthreads();
@@ -118,34 +132,31 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #ifdef MUSE_PHASE_CLOCKS
     long long pc[6] = {0, 0, 0, 0, 0, 0};
 #endif
-    float bnext = beta[ent0 + L];
-    auto issue_kappa = [&](int jt_) {                       // issuer: the two kappa tiles of cluster tile jt_
-      tc::mbar_expect_tx(&bar_full, 2 * kTile);
-      const int row = (int)(ent0 + (size_t)jt_ * TJ);
-      tc::tma_load_2d(sm + oHi, &tm_khi, 0, row, &bar_full); tc::tma_load_2d(sm + oHi + TJ * 128, &tm_khi, 64, row, &bar_full);
-      tc::tma_load_2d(sm + oLo, &tm_klo, 0, row, &bar_full); tc::tma_load_2d(sm + oLo + TJ * 128, &tm_klo, 64, row, &bar_full);
-    };
-    auto issue_nu = [&](int jt_) {                          // issuer: its nu tile
-      tc::mbar_expect_tx(&bar_nu, kTile);
-      const int row = (int)(ent0 + (size_t)jt_ * TJ);
-      tc::tma_load_2d(sm + oNu, &tm_nu, 0, row, &bar_nu); tc::tma_load_2d(sm + oNu + TJ * 128, &tm_nu, 64, row, &bar_nu);
-    };
-    const bool later_sweep = s0 > p0;                       // gradients of earlier sweeps are already stored: add to them
-    if (tid == ISSUER) {
-      if (later_sweep) tc::tma_store_wait_all();
-      issue_kappa(0);
-      issue_nu(0);
+    // L and delta of this warpgroup's 32 rows stay in registers for the whole sweep
+    static_assert(NP == 1, "one pass per sweep");
+    float Lc[32], dc[32];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const float4 a = *reinterpret_cast<const float4*>(Ls + 32 * (wg & 1) + 4 * k), b = *reinterpret_cast<const float4*>(ds + 32 * (wg & 1) + 4 * k);
+      Lc[4 * k] = a.x; Lc[4 * k + 1] = a.y; Lc[4 * k + 2] = a.z; Lc[4 * k + 3] = a.w;
+      dc[4 * k] = b.x; dc[4 * k + 1] = b.y; dc[4 * k + 2] = b.z; dc[4 * k + 3] = b.w;
     }
-    if (later_sweep) __syncthreads();
+    float bnext = beta[ent0 + L];
+    const bool later_sweep = s0 > p0;                       // gradients of earlier sweeps are already stored: add to them
+    if (later_sweep) {
+      if (tid == ISSUER) tc::tma_store_wait_all();
+      __syncthreads();
+    }
     for (int jt = 0; jt < NJ && ok; ++jt) {
       const int j = jt * TJ + L;
 #ifdef MUSE_PHASE_CLOCKS
       long long k0_ = clock64(), k1_ = 0, k2_ = 0, k3_ = 0, k4_ = 0;
 #endif
       const float bj = bnext;                               // loaded one tile ahead
-      const float sig2 = dm.sigma * kLog2e, bj2 = bj * kLog2e;
+      const bool alive = bj != -INFINITY;                   // an empty cluster has beta = mu = -inf
+      const float sig2 = dm.sigma * kLog2e, bj2 = alive ? bj * kLog2e : 0.f;
       if (jt + 1 < NJ) bnext = beta[ent0 + j + TJ];
-      float gsum = 0.f, dsum = 0.f;
+      float gsum = 0.f, gt2 = 0.f, pdp = 0.f;
       const float mu1 = 1.f + mu[ent0 + j];                               // 1 + accumulated log-mass of cluster j
       for (int p = 0; p < np && ok; ++p) {
         const uint32_t aQ = tc::smem_u32(sm + oQ + p * kRows), aDO = tc::smem_u32(sm + oDO + p * kRows);
@@ -190,34 +201,22 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
           if (p == 0 && tid == 0 && blockIdx.x == 5 && blockIdx.y == 3 && blockIdx.z == 0 && jt == 3) status[32] = (int)(clock64() - k1_);
 #endif
           uint32_t pw[16], gw[16];
-          // per-row L, delta and retrieved-cluster bits: vector loads ahead of the arithmetic loop
-          float Lc[32], dc[32];
-          uint32_t mk[32];
-          const int rb = p * NR + 32 * wg;
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const float4 a = *reinterpret_cast<const float4*>(Ls + rb + 4 * k), b = *reinterpret_cast<const float4*>(ds + rb + 4 * k);
-            const uint4 w = *reinterpret_cast<const uint4*>(smask + (j >> 5) * (NP * NR) + rb + 4 * k);
-            Lc[4 * k] = a.x; Lc[4 * k + 1] = a.y; Lc[4 * k + 2] = a.z; Lc[4 * k + 3] = a.w;
-            dc[4 * k] = b.x; dc[4 * k + 1] = b.y; dc[4 * k + 2] = b.z; dc[4 * k + 3] = b.w;
-            mk[4 * k] = w.x; mk[4 * k + 1] = w.y; mk[4 * k + 2] = w.z; mk[4 * k + 3] = w.w;
-          }
-          const bool alive = bj != -INFINITY;
+          // bit r of `near`: row r of this warpgroup's 32 is not in the far set of cluster j (retrieved,
+          // past the end of the segment, or the cluster is empty)
+          const int nv = ns - (p * NR + 32 * wg);
+          const uint32_t near = alive ? (smask[2 * j + wg] | (nv >= 32 ? 0u : nv <= 0 ? 0xffffffffu : 0xffffffffu << nv)) : 0xffffffffu;
 #pragma unroll
           for (int c = 0; c < 32; c += 2) {
             float pv[2], gv[2];
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-              const bool far = alive && rb + c + h < ns && !((mk[c + h] >> (j & 31)) & 1u);
               const float t2 = fmaf(s[c + h], sig2, bj2);                 // Eq. 6 score in log2 units
               const float e = fast_exp2(t2 - Lc[c + h]);
-              pv[h] = far ? e : 0.f;
+              pv[h] = (near >> (c + h)) & 1u ? 0.f : e;
               gv[h] = pv[h] * (dp[c + h] - dc[c + h]);
               gsum += gv[h];
-              // dS = sum_r g (1 + mu - score) - sum_r p (dO.nu): the same quantity as
-              // sum_r g - dkappa.kappa - dnu.nu, without the two row dot products
-              dsum = fmaf(gv[h], far ? fmaf(-t2, 0.6931471805599453f, mu1) : 0.f, dsum);    // (an empty cluster has mu = -inf)
-              dsum = fmaf(-pv[h], dp[c + h], dsum);
+              gt2 = fmaf(gv[h], t2, gt2);
+              pdp = fmaf(pv[h], dp[c + h], pdp);
             }
             __nv_bfloat162 a = __floats2bfloat162_rn(pv[0], pv[1]), b = __floats2bfloat162_rn(gv[0], gv[1]);
             pw[c >> 1] = *reinterpret_cast<uint32_t*>(&a);
@@ -282,7 +281,9 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       // ---- tile read-out: warpgroup 0 -> dnu, warpgroup 1 -> dkappa; both need sum_r g
       float gtot = 0.f;
       if (cw) {
-        part[wg][L] = gsum; dsid[wg][L] = dsum;
+        // dS = sum_r g (1 + mu - score) - sum_r p (dO.nu): the same quantity as
+        // sum_r g - dkappa.kappa - dnu.nu, without the two row dot products
+        part[wg][L] = gsum; dsid[wg][L] = alive ? fmaf(mu1, gsum, fmaf(-0.6931471805599453f, gt2, -pdp)) : 0.f;
         tc::named_bar_sync(1, CW);                          // the issuer is still waiting for the dq products
         gtot = part[0][L] + part[1][L];
       }
@@ -356,7 +357,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #pragma unroll
           for (int r = 0; r < 32; ++r) {
             const int rr = p * NR + c0 + r;
-            if (rr < ns) dQacc[((size_t)pq * dm.N + rows[rr]) * D + L] += dm.sigma * v[r];
+            if (rr < ns) atomicAdd(dQacc + ((size_t)pq * dm.N + rows[rr]) * D + L, dm.sigma * v[r]);   // (result unused: no round trip)
           }
         }
       }
@@ -365,7 +366,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   }
   tc::fence_before_sync();
   __syncthreads();
-  if (tid == ISSUER) tc::tma_store_wait_all();
+  if (tid == ISSUER) tc::tma_store_wait_read();             // the staging tiles must outlive the stores' reads only
   if (warp == 0) tc::tmem_dealloc(tbase, 512);
   if (!ok && tid == 0) atomicExch(status, 4);
 }
