@@ -287,17 +287,18 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
         tc::named_bar_sync(1, CW);                          // the issuer is still waiting for the dq products
         gtot = part[0][L] + part[1][L];
       }
+#ifdef MUSE_PHASE_CLOCKS
+      const bool rec_ = (tid == 0 || tid == 128) && blockIdx.x == 5 && blockIdx.y == 3 && blockIdx.z == 0 && jt == 3;
+      if (rec_) status[34 + 3 * wg] = (int)(clock64() - k3_);
+#endif
       // gradient entry: [plane][i][j] like the summaries, or [plane][j][i] so that the key-side
       // pass finds the 128 query clusters of one key cluster in one contiguous tile
       const size_t gent = grad_by_key_cluster ? (((size_t)pq * dm.SB + pl) * Ck + j) * dm.Cq + i : ent0 + j;
+      // 16 dims of this thread's row: scale, round, into its own row of the staging tile (which then
+      // leaves as one TMA box)
+      auto emit = [&](const float (&v)[16], int d0) {
 #pragma unroll
-      for (int d0 = 0; cw && d0 < D; d0 += 32) {
-        float v[32];
-        tc::tmem_ld32(tlane + (wg == 0 ? cDNU : cDKA) + d0, v);
-        // the second half of the dkappa staging is the G tile, which the dq products read
-        if (wg == 1 && d0 == 64 && !tc::mbar_wait(&bar3, ph3 ^ 1)) ok = false;
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
+        for (int ch = 0; ch < 2; ++ch) {
           const int d = d0 + 8 * ch;
           float x[8];
           if (wg == 0) {
@@ -309,25 +310,47 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #pragma unroll
             for (int e = 0; e < 8; ++e) x[e] = dm.sigma * (v[8 * ch + e] - gtot * qv[e]);
           }
-          uint32_t w[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) { __nv_bfloat162 b2 = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]); w[e] = *reinterpret_cast<uint32_t*>(&b2); }
-          // into this thread's own row of the staging tile, which then leaves as one TMA box
-          const int kb = d >> 6, c = (d & 63) >> 3;
           if (later_sweep) {
             const bf16* old = (wg == 0 ? dnu : dkappa) + gent * D + d;
             const float4 o0 = ld4(old), o1 = ld4(old + 4);
             x[0] += o0.x; x[1] += o0.y; x[2] += o0.z; x[3] += o0.w; x[4] += o1.x; x[5] += o1.y; x[6] += o1.z; x[7] += o1.w;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) { __nv_bfloat162 b2 = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]); w[e] = *reinterpret_cast<uint32_t*>(&b2); }
           }
+          uint32_t w[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) { __nv_bfloat162 b2 = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]); w[e] = *reinterpret_cast<uint32_t*>(&b2); }
+          const int kb = d >> 6, c = (d & 63) >> 3;
           *reinterpret_cast<uint4*>(sm + (wg == 0 ? oStN : oStK) + kb * TJ * 128 + tc::sw128_off(L, c)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
+      };
+      if (cw) {
+        // two 16-column loads stay in flight while the two before them are converted
+        const uint32_t tsrc = tlane + (wg == 0 ? cDNU : cDKA);
+        float va[16], vb[16], vc[16], vd[16];
+        tc::tmem_ld16_issue(tsrc, va); tc::tmem_ld16_issue(tsrc + 16, vb);
+        tc::tmem_ld_wait(); tc::tmem_ld_use16(va); tc::tmem_ld_use16(vb);
+        tc::tmem_ld16_issue(tsrc + 32, vc); tc::tmem_ld16_issue(tsrc + 48, vd);
+        emit(va, 0); emit(vb, 16);
+        tc::tmem_ld_wait(); tc::tmem_ld_use16(vc); tc::tmem_ld_use16(vd);
+        tc::tmem_ld16_issue(tsrc + 64, va); tc::tmem_ld16_issue(tsrc + 80, vb);
+        emit(vc, 32); emit(vd, 48);
+        tc::tmem_ld_wait(); tc::tmem_ld_use16(va); tc::tmem_ld_use16(vb);
+        tc::tmem_ld16_issue(tsrc + 96, vc); tc::tmem_ld16_issue(tsrc + 112, vd);
+        // the second half of the dkappa staging is the G tile, which the dq products read
+        if (wg == 1 && !tc::mbar_wait(&bar3, ph3 ^ 1)) ok = false;
+        emit(va, 64); emit(vb, 80);
+        tc::tmem_ld_wait(); tc::tmem_ld_use16(vc); tc::tmem_ld_use16(vd);
+        emit(vc, 96); emit(vd, 112);
       }
+#ifdef MUSE_PHASE_CLOCKS
+      if (rec_) status[35 + 3 * wg] = (int)(clock64() - k3_);
+#endif
       // the two gradient tiles leave by TMA: 128 rows of 256 bytes each, Cq entries apart in the
       // [plane][j][i] layout (adjacent in the [plane][i][j] one)
       tc::fence_async_smem();
       __syncthreads();
+#ifdef MUSE_PHASE_CLOCKS
+      if (rec_) status[36 + 3 * wg] = (int)(clock64() - k3_);
+#endif
       if (tid == ISSUER && ok) {
         const int c1 = grad_by_key_cluster ? i : 0;
         const int c2 = grad_by_key_cluster ? (pq * dm.SB + pl) * Ck + jt * TJ : (int)(ent0 + (size_t)jt * TJ);
