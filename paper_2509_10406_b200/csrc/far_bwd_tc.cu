@@ -62,6 +62,10 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   const int i = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z;
   const int blk = dm.causal ? pl + 1 : 0, Ck = dm.Ck, NJ = Ck / TJ, MW = Ck >> 5, m = dm.m;
   const int tid = threadIdx.x, warp = tid >> 5, wg = tid >> 7, L = tid & 127;
+#ifdef MUSE_PHASE_CLOCKS
+  const long long t_in_ = clock64();
+  long long t_loop_ = 0, t_end_ = 0;
+#endif
   const int32_t* oq = off_q + (size_t)pq * (dm.S * dm.Cq + 1) + (size_t)blk * dm.Cq + i;
   const int p0 = oq[0], p1 = oq[1];
   if (p0 >= p1) return;
@@ -147,6 +151,9 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       if (tid == ISSUER) tc::tma_store_wait_all();
       __syncthreads();
     }
+#ifdef MUSE_PHASE_CLOCKS
+    t_loop_ = clock64();
+#endif
     for (int jt = 0; jt < NJ && ok; ++jt) {
       const int j = jt * TJ + L;
 #ifdef MUSE_PHASE_CLOCKS
@@ -294,52 +301,38 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       // gradient entry: [plane][i][j] like the summaries, or [plane][j][i] so that the key-side
       // pass finds the 128 query clusters of one key cluster in one contiguous tile
       const size_t gent = grad_by_key_cluster ? (((size_t)pq * dm.SB + pl) * Ck + j) * dm.Cq + i : ent0 + j;
-      // 16 dims of this thread's row: scale, round, into its own row of the staging tile (which then
-      // leaves as one TMA box)
-      auto emit = [&](const float (&v)[16], int d0) {
+      // this thread's row, 32 dims per step: row = scale (acc - gq qbar_i) with (scale, gq) = (1, 0) for dnu and
+      // (sigma, sum_r g) for dkappa, rounded into its own row of the staging tile (which then leaves as one
+      // TMA box).  The next 32 columns travel from TMEM while these are converted.
+      if (cw) {
+        const uint32_t tsrc = tlane + (wg == 0 ? cDNU : cDKA);
+        unsigned char* stg = sm + (wg == 0 ? oStN : oStK) + L * 128;
+        const float sc = wg == 0 ? 1.f : dm.sigma, gq = wg == 0 ? 0.f : gtot;
+        float va[16], vb[16];
+        tc::tmem_ld16_issue(tsrc, va); tc::tmem_ld16_issue(tsrc + 16, vb);
+#pragma unroll 1
+        for (int u = 0; u < D / 32; ++u) {
+          tc::tmem_ld_wait(); tc::tmem_ld_use16(va); tc::tmem_ld_use16(vb);
+          float x[32];
 #pragma unroll
-        for (int ch = 0; ch < 2; ++ch) {
-          const int d = d0 + 8 * ch;
-          float x[8];
-          if (wg == 0) {
+          for (int e = 0; e < 16; ++e) { x[e] = va[e]; x[16 + e] = vb[e]; }
+          if (u + 1 < D / 32) { tc::tmem_ld16_issue(tsrc + 32 * (u + 1), va); tc::tmem_ld16_issue(tsrc + 32 * (u + 1) + 16, vb); }
+          // the second half of the dkappa staging is the G tile, which the dq products read
+          if (u == 2 && wg == 1 && !tc::mbar_wait(&bar3, ph3 ^ 1)) ok = false;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) x[e] = v[8 * ch + e];
-          } else {
+          for (int ch = 0; ch < 4; ++ch) {
+            const int d = 32 * u + 8 * ch;
             const float4 q0 = *reinterpret_cast<const float4*>(qb + d), q1 = *reinterpret_cast<const float4*>(qb + d + 4);
             const float qv[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
+            uint32_t w[4];
 #pragma unroll
-            for (int e = 0; e < 8; ++e) x[e] = dm.sigma * (v[8 * ch + e] - gtot * qv[e]);
+            for (int e = 0; e < 4; ++e) {
+              __nv_bfloat162 b2 = __floats2bfloat162_rn(sc * fmaf(-gq, qv[2 * e], x[8 * ch + 2 * e]), sc * fmaf(-gq, qv[2 * e + 1], x[8 * ch + 2 * e + 1]));
+              w[e] = *reinterpret_cast<uint32_t*>(&b2);
+            }
+            *reinterpret_cast<uint4*>(stg + (d >> 6) * (TJ * 128) + (((((d & 63) >> 3)) ^ (L & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
           }
-          if (later_sweep) {
-            const bf16* old = (wg == 0 ? dnu : dkappa) + gent * D + d;
-            const float4 o0 = ld4(old), o1 = ld4(old + 4);
-            x[0] += o0.x; x[1] += o0.y; x[2] += o0.z; x[3] += o0.w; x[4] += o1.x; x[5] += o1.y; x[6] += o1.z; x[7] += o1.w;
-          }
-          uint32_t w[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) { __nv_bfloat162 b2 = __floats2bfloat162_rn(x[2 * e], x[2 * e + 1]); w[e] = *reinterpret_cast<uint32_t*>(&b2); }
-          const int kb = d >> 6, c = (d & 63) >> 3;
-          *reinterpret_cast<uint4*>(sm + (wg == 0 ? oStN : oStK) + kb * TJ * 128 + tc::sw128_off(L, c)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-      };
-      if (cw) {
-        // two 16-column loads stay in flight while the two before them are converted
-        const uint32_t tsrc = tlane + (wg == 0 ? cDNU : cDKA);
-        float va[16], vb[16], vc[16], vd[16];
-        tc::tmem_ld16_issue(tsrc, va); tc::tmem_ld16_issue(tsrc + 16, vb);
-        tc::tmem_ld_wait(); tc::tmem_ld_use16(va); tc::tmem_ld_use16(vb);
-        tc::tmem_ld16_issue(tsrc + 32, vc); tc::tmem_ld16_issue(tsrc + 48, vd);
-        emit(va, 0); emit(vb, 16);
-        tc::tmem_ld_wait(); tc::tmem_ld_use16(vc); tc::tmem_ld_use16(vd);
-        tc::tmem_ld16_issue(tsrc + 64, va); tc::tmem_ld16_issue(tsrc + 80, vb);
-        emit(vc, 32); emit(vd, 48);
-        tc::tmem_ld_wait(); tc::tmem_ld_use16(va); tc::tmem_ld_use16(vb);
-        tc::tmem_ld16_issue(tsrc + 96, vc); tc::tmem_ld16_issue(tsrc + 112, vd);
-        // the second half of the dkappa staging is the G tile, which the dq products read
-        if (wg == 1 && !tc::mbar_wait(&bar3, ph3 ^ 1)) ok = false;
-        emit(va, 64); emit(vb, 80);
-        tc::tmem_ld_wait(); tc::tmem_ld_use16(vc); tc::tmem_ld_use16(vd);
-        emit(vc, 96); emit(vd, 112);
       }
 #ifdef MUSE_PHASE_CLOCKS
       if (rec_) status[35 + 3 * wg] = (int)(clock64() - k3_);
@@ -354,8 +347,13 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       if (tid == ISSUER && ok) {
         const int c1 = grad_by_key_cluster ? i : 0;
         const int c2 = grad_by_key_cluster ? (pq * dm.SB + pl) * Ck + jt * TJ : (int)(ent0 + (size_t)jt * TJ);
-        tc::tma_store_3d(&tm_gnu, sm + oStN, 0, c1, c2); tc::tma_store_3d(&tm_gnu, sm + oStN + TJ * 128, 64, c1, c2);
-        tc::tma_store_3d(&tm_gka, sm + oStK, 0, c1, c2); tc::tma_store_3d(&tm_gka, sm + oStK + TJ * 128, 64, c1, c2);
+        if (!later_sweep) {
+          tc::tma_store_3d(&tm_gnu, sm + oStN, 0, c1, c2); tc::tma_store_3d(&tm_gnu, sm + oStN + TJ * 128, 64, c1, c2);
+          tc::tma_store_3d(&tm_gka, sm + oStK, 0, c1, c2); tc::tma_store_3d(&tm_gka, sm + oStK + TJ * 128, 64, c1, c2);
+        } else {                              // a further sweep of a long segment adds to the stored rows
+          tc::tma_reduce_add_3d(&tm_gnu, sm + oStN, 0, c1, c2); tc::tma_reduce_add_3d(&tm_gnu, sm + oStN + TJ * 128, 64, c1, c2);
+          tc::tma_reduce_add_3d(&tm_gka, sm + oStK, 0, c1, c2); tc::tma_reduce_add_3d(&tm_gka, sm + oStK + TJ * 128, 64, c1, c2);
+        }
         tc::tma_store_commit();
       }
       tc::fence_before_sync();
@@ -368,6 +366,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #ifdef MUSE_PHASE_CLOCKS
     if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 3 && blockIdx.z == 0 && s0 == p0)
       for (int k = 0; k < 6; ++k) status[24 + k] = (int)pc[k];
+    t_end_ = clock64();
 #endif
     // ---- dq: warpgroup p reads pass p (thread = output dim), adds into the fp32 accumulator
     if (cw && !tc::mbar_wait(&bar3, ph3 ^ 1)) ok = false;     // the last tile's dq products
@@ -392,6 +391,11 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   if (tid == ISSUER) tc::tma_store_wait_read();             // the staging tiles must outlive the stores' reads only
   if (warp == 0) tc::tmem_dealloc(tbase, 512);
   if (!ok && tid == 0) atomicExch(status, 4);
+#ifdef MUSE_PHASE_CLOCKS
+  if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 3 && blockIdx.z == 0) {
+    status[56] = (int)(t_loop_ - t_in_); status[57] = (int)(t_end_ - t_loop_); status[58] = (int)(clock64() - t_end_);
+  }
+#endif
 }
 
 bool far_bwd_tc_supported(const Dims& d, int dtype) {
