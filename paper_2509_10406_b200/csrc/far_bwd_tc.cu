@@ -4,8 +4,8 @@
 // takes further sweeps that add to the stored gradients).  Per cluster tile, with L the merged log-sum-exp and delta = dO.O:
 //   S^T   = (kappa_hi + kappa_lo) Q^T,  dPnu^T = nu dO^T                      (tcgen05, TMA-fed tiles)
 //   p     = exp(sigma S + beta - L) on the far set,  g = p (dPnu - delta)      (one thread per cluster)
-//   dnu  += p dO,   dkappa_raw += g Q,   dq^T += kappa^T g                     (tcgen05)
-//   dkappa = sigma (dkappa_raw - (sum_r g) qbar_i)
+//   dnu  += p dO,   dkappa_raw += (sigma g) Q,   dq^T += kappa^T (sigma g)     (tcgen05; the G tile carries sigma)
+//   dkappa = dkappa_raw - sigma (sum_r g) qbar_i
 //   dS = sum_r g - dkappa.kappa - dnu.nu = sum_r g (1 + mu - score) - sum_r p dPnu   (no row dot products)
 // dkappa and dnu are stored as bf16 rows for the key-side pass, dS as fp32.
 #include <cuda.h>
@@ -225,7 +225,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
               gt2 = fmaf(gv[h], t2, gt2);
               pdp = fmaf(pv[h], dp[c + h], pdp);
             }
-            __nv_bfloat162 a = __floats2bfloat162_rn(pv[0], pv[1]), b = __floats2bfloat162_rn(gv[0], gv[1]);
+            __nv_bfloat162 a = __floats2bfloat162_rn(pv[0], pv[1]), b = __floats2bfloat162_rn(dm.sigma * gv[0], dm.sigma * gv[1]);
             pw[c >> 1] = *reinterpret_cast<uint32_t*>(&a);
             gw[c >> 1] = *reinterpret_cast<uint32_t*>(&b);
           }
@@ -301,33 +301,34 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       // gradient entry: [plane][i][j] like the summaries, or [plane][j][i] so that the key-side
       // pass finds the 128 query clusters of one key cluster in one contiguous tile
       const size_t gent = grad_by_key_cluster ? (((size_t)pq * dm.SB + pl) * Ck + j) * dm.Cq + i : ent0 + j;
-      // this thread's row, 32 dims per step: row = scale (acc - gq qbar_i) with (scale, gq) = (1, 0) for dnu and
-      // (sigma, sum_r g) for dkappa, rounded into its own row of the staging tile (which then leaves as one
-      // TMA box).  The next 32 columns travel from TMEM while these are converted.
+      // this thread's row, 32 dims per step, rounded into its own row of the staging tile (which then leaves
+      // as one TMA box).  The G tile carried sigma, so dkappa = acc - (sigma sum_r g) qbar_i.  (Few instructions
+      // per element matter more here than overlapping the TMEM loads: eight warps share the issue slots.)
       if (cw) {
         const uint32_t tsrc = tlane + (wg == 0 ? cDNU : cDKA);
         unsigned char* stg = sm + (wg == 0 ? oStN : oStK) + L * 128;
-        const float sc = wg == 0 ? 1.f : dm.sigma, gq = wg == 0 ? 0.f : gtot;
-        float va[16], vb[16];
-        tc::tmem_ld16_issue(tsrc, va); tc::tmem_ld16_issue(tsrc + 16, vb);
+        const float gq = -dm.sigma * gtot;
 #pragma unroll 1
         for (int u = 0; u < D / 32; ++u) {
-          tc::tmem_ld_wait(); tc::tmem_ld_use16(va); tc::tmem_ld_use16(vb);
           float x[32];
-#pragma unroll
-          for (int e = 0; e < 16; ++e) { x[e] = va[e]; x[16 + e] = vb[e]; }
-          if (u + 1 < D / 32) { tc::tmem_ld16_issue(tsrc + 32 * (u + 1), va); tc::tmem_ld16_issue(tsrc + 32 * (u + 1) + 16, vb); }
+          tc::tmem_ld32(tsrc + 32 * u, x);
           // the second half of the dkappa staging is the G tile, which the dq products read
           if (u == 2 && wg == 1 && !tc::mbar_wait(&bar3, ph3 ^ 1)) ok = false;
+          if (wg == 1) {
+#pragma unroll
+            for (int ch = 0; ch < 8; ++ch) {
+              const float4 q = *reinterpret_cast<const float4*>(qb + 32 * u + 4 * ch);
+              x[4 * ch] = fmaf(gq, q.x, x[4 * ch]); x[4 * ch + 1] = fmaf(gq, q.y, x[4 * ch + 1]);
+              x[4 * ch + 2] = fmaf(gq, q.z, x[4 * ch + 2]); x[4 * ch + 3] = fmaf(gq, q.w, x[4 * ch + 3]);
+            }
+          }
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
             const int d = 32 * u + 8 * ch;
-            const float4 q0 = *reinterpret_cast<const float4*>(qb + d), q1 = *reinterpret_cast<const float4*>(qb + d + 4);
-            const float qv[8] = {q0.x, q0.y, q0.z, q0.w, q1.x, q1.y, q1.z, q1.w};
             uint32_t w[4];
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              __nv_bfloat162 b2 = __floats2bfloat162_rn(sc * fmaf(-gq, qv[2 * e], x[8 * ch + 2 * e]), sc * fmaf(-gq, qv[2 * e + 1], x[8 * ch + 2 * e + 1]));
+              __nv_bfloat162 b2 = __floats2bfloat162_rn(x[8 * ch + 2 * e], x[8 * ch + 2 * e + 1]);
               w[e] = *reinterpret_cast<uint32_t*>(&b2);
             }
             *reinterpret_cast<uint4*>(stg + (d >> 6) * (TJ * 128) + (((((d & 63) >> 3)) ^ (L & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -379,7 +380,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #pragma unroll
           for (int r = 0; r < 32; ++r) {
             const int rr = p * NR + c0 + r;
-            if (rr < ns) atomicAdd(dQacc + ((size_t)pq * dm.N + rows[rr]) * D + L, dm.sigma * v[r]);   // (result unused: no round trip)
+            if (rr < ns) atomicAdd(dQacc + ((size_t)pq * dm.N + rows[rr]) * D + L, v[r]);   // (result unused: no round trip)
           }
         }
       }
