@@ -68,7 +68,20 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #endif
   const int32_t* oq = off_q + (size_t)pq * (dm.S * dm.Cq + 1) + (size_t)blk * dm.Cq + i;
   const int p0 = oq[0], p1 = oq[1];
-  if (p0 >= p1) return;
+  if (p0 >= p1) {
+    // An empty segment: its gradient rows are zeros.  The key-side tensor-core pass (the reader of the
+    // [plane][j][i] layout) takes whole tiles of rows without looking at which segments exist.
+    if (grad_by_key_cluster) {
+      const size_t row0 = ((size_t)pq * dm.SB + pl) * Ck;
+      for (int e = tid; e < Ck * (D / 8); e += blockDim.x) {
+        const size_t at = ((row0 + (e >> 4)) * dm.Cq + i) * D + (e & 15) * 8;
+        *reinterpret_cast<uint4*>(dkappa + at) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(dnu + at) = make_uint4(0u, 0u, 0u, 0u);
+      }
+      for (int j = tid; j < Ck; j += blockDim.x) dS[(row0 + j) * dm.Cq + i] = 0.f;
+    }
+    return;
+  }
   unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
   uint32_t* smask = reinterpret_cast<uint32_t*>(sm + oMask);
   const size_t ent0 = (((size_t)pq * dm.SB + pl) * dm.Cq + i) * Ck;

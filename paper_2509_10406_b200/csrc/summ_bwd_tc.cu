@@ -140,7 +140,11 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
       tc::fence_after_sync();
       PCLK(0)
       float lg[32];
-      if (cw) tc::tmem_ld32(tlane + cL + 32 * wg, lg);            // this thread's logits: row i, keys 32 wg .. 32 wg + 31
+      if (cw) {                                                   // this thread's logits: row i, keys 32 wg .. 32 wg + 31 (log2 units)
+        tc::tmem_ld32(tlane + cL + 32 * wg, lg);
+#pragma unroll
+        for (int c = 0; c < 32; ++c) lg[c] *= 1.4426950408889634f;
+      }
       // per-plane scalars, loaded one plane ahead
       auto ent_of = [&](int pl) { return (((size_t)pq * dm.SB + pl) * dm.Cq + ic) * dm.Ck + j; };        // summaries: [plane][i][j]
       auto gent_of = [&](int pl) { return (((size_t)pq * dm.SB + pl) * dm.Ck + j) * dm.Cq + ic; };      // gradients: [plane][j][i]
@@ -150,34 +154,16 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         const int buf = k & 1;
         const int nk = min(NU, ok_[pl + 1] - c0);
         const bool live = (livemask >> pl) & 1u;
-        const float mu_i = mu_n, dS_i = dS_n;
-        if (k > 0) {                                      // the MMAs of the previous plane are done with the other buffer and with W / Wc
-          if (!tc::mbar_wait(&bar2, ph2)) ok = false;
-          ph2 ^= 1;
-          tc::fence_after_sync();
-        }
-        PCLK(1)
-        if (tid == ISSUER && pl + 1 < dm.SB && ok) issue_grad(pl + 1, buf ^ 1);
-        if (pl + 1 < dm.SB && ((livemask >> (pl + 1)) & 1u)) { mu_n = mu[ent_of(pl + 1)]; dS_n = dS[gent_of(pl + 1)]; }
-        if (!tc::mbar_wait(&bar_g[buf], ph_g[buf])) ok = false;
-        ph_g[buf] ^= 1;
-        PCLK(2)
+        const float mu_i = mu_n * 1.4426950408889634f, dS_i = dS_n;
         const int oDka = buf ? oQlo : oDka0, oDnu = buf ? oDnu1 : oDnu0;
-        // rows of query clusters whose segment is empty (or beyond Cq) were never written: clear them
-        if (cw && !live) {
-#pragma unroll
-          for (int c8 = 0; c8 < D / 16; ++c8) {
-            const int ck = wg * (D / 16) + c8;
-            const uint32_t off = (ck >> 3) * TI * 128 + tc::sw128_off(L, ck & 7);
-            *reinterpret_cast<uint4*>(sm + oDka + off) = make_uint4(0u, 0u, 0u, 0u);
-            *reinterpret_cast<uint4*>(sm + oDnu + off) = make_uint4(0u, 0u, 0u, 0u);
-          }
-        }
-        tc::fence_async_smem();
-        tc::fence_before_sync();
-        __syncthreads();
         const uint32_t aDka = tc::smem_u32(sm + oDka), aDnu = tc::smem_u32(sm + oDnu);
+        if (pl + 1 < dm.SB && ((livemask >> (pl + 1)) & 1u)) { mu_n = mu[ent_of(pl + 1)]; dS_n = dS[gent_of(pl + 1)]; }
+        // The far-field pass wrote every row of the gradient tensors (zeros for an empty segment), so the
+        // tiles go to the tensor cores as they land.  The D-contractions of this plane do not depend on the
+        // previous plane's i-contractions: they are issued first, and only the W / Wc tiles and the other
+        // gradient buffer wait for those.
         if (tid == ISSUER) {
+          if (!tc::mbar_wait(&bar_g[buf], ph_g[buf])) ok = false;
           tc::fence_after_sync();
           const uint32_t idesc = tc::idesc_bf16(TI, NU, 0, 0);
 #pragma unroll
@@ -189,9 +175,12 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
             tc::mma_bf16_ss(tbase + cX2, tc::smem_desc_sw128(aDnu + (ks / 4) * TI * 128 + (ks % 4) * 32, 16, 1024),
                             tc::smem_desc_sw128(aV + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
           tc::mma_commit(&bar1);
+          if (k > 0 && !tc::mbar_wait(&bar2, ph2)) ok = false;      // the previous plane's MMAs are done with the other buffer
+          if (pl + 1 < dm.SB && ok) issue_grad(pl + 1, buf ^ 1);
         }
-        __syncwarp();
-        if (!tc::mbar_wait(&bar1, ph1)) ok = false;
+        ph_g[buf] ^= 1;
+        PCLK(1)
+        if (cw && !tc::mbar_wait(&bar1, ph1)) ok = false;
         ph1 ^= 1;
         tc::fence_after_sync();
         PCLK(3)
@@ -203,17 +192,19 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
 #pragma unroll
           for (int c = 0; c < 32; c += 2) {
             float w0 = 0.f, w1 = 0.f, c0_ = 0.f, c1_ = 0.f;
-            if (live && 32 * wg + c < nk) { w0 = __expf(lg[c] - mu_i); c0_ = w0 * (dS_i + x1[c] + x2[c]); }
-            if (live && 32 * wg + c + 1 < nk) { w1 = __expf(lg[c + 1] - mu_i); c1_ = w1 * (dS_i + x1[c + 1] + x2[c + 1]); }
+            if (live && 32 * wg + c < nk) { w0 = tc::fast_exp2(lg[c] - mu_i); c0_ = w0 * (dS_i + x1[c] + x2[c]); }
+            if (live && 32 * wg + c + 1 < nk) { w1 = tc::fast_exp2(lg[c + 1] - mu_i); c1_ = w1 * (dS_i + x1[c + 1] + x2[c + 1]); }
             __nv_bfloat162 a = __floats2bfloat162_rn(w0, w1), b = __floats2bfloat162_rn(c0_, c1_);
             ww[c >> 1] = *reinterpret_cast<uint32_t*>(&a); wc[c >> 1] = *reinterpret_cast<uint32_t*>(&b);
           }
+          if (k > 0 && !tc::mbar_wait(&bar2, ph2)) ok = false;      // the previous plane's MMAs have read W / Wc
 #pragma unroll
           for (int ch = 0; ch < 4; ++ch) {
             *reinterpret_cast<uint4*>(sm + oW + tc::sw128_off(L, 4 * wg + ch)) = make_uint4(ww[4 * ch], ww[4 * ch + 1], ww[4 * ch + 2], ww[4 * ch + 3]);
             *reinterpret_cast<uint4*>(sm + oWc + tc::sw128_off(L, 4 * wg + ch)) = make_uint4(wc[4 * ch], wc[4 * ch + 1], wc[4 * ch + 2], wc[4 * ch + 3]);
           }
         }
+        if (k > 0) ph2 ^= 1;
         tc::fence_async_smem();
         tc::fence_before_sync();
         __syncthreads();
@@ -261,8 +252,8 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         for (int u = 0; u < 32; ++u) {
           if (32 * wg + u < nkc) {
             const size_t at = ((size_t)pq * dm.N + c0 + 32 * wg + u) * D + L;
-            dK_perm[at] += a[u];
-            dV_perm[at] += b[u];
+            atomicAdd(dK_perm + at, a[u]);                 // (result unused: no round trip; one CTA owns the element)
+            atomicAdd(dV_perm + at, b[u]);
           }
         }
       }
@@ -273,7 +264,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tbase, 512);
 #ifdef MUSE_PHASE_CLOCKS
-  if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 0) for (int k = 0; k < 8; ++k) status[56 + k] = 0 * (int)pc[k];
+  if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 0) for (int k = 0; k < 8; ++k) status[56 + k] = (int)pc[k];
 #endif
   if (!ok && tid == 0) atomicExch(status, 5);
 }
