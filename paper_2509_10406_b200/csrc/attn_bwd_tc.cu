@@ -707,20 +707,32 @@ k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
 //   S = Q K^T, dP = dO V^T  ->  P = exp(sigma S - L), G = P (dP - delta)   (one thread per pair row)
 //   dQ   += G K                     [pairs][D]   written per pair as a bf16 row
 //   dV^T += dO^T P,  dK^T += Q^T G  [D][keys]    accumulated in TMEM over all tiles and planes
-// Q and dO rows are gathered once for all three products, one tile ahead (registers), their pair
-// ids two tiles ahead, across plane boundaries.  The CTA owns the cluster's keys for its head, so
-// dK and dV leave with plain coalesced read-modify-writes (thread = output dim).
+// Eight warps do the arithmetic; lane 0 of a ninth warp issues every MMA, so that the first
+// products of the next chunk (or tile) queue behind the second batch of the current one.  The Q and
+// dO rows of a tile are gathered once for all three products, one tile ahead, by asynchronous
+// 16-byte copies straight into the other half of a double buffer; pair ids run two tiles ahead,
+// across plane boundaries.  The CTA owns the cluster's keys for its head (or shares them with up
+// to three others): dK and dV leave as fire-and-forget adds, thread = output dim.
 // ================================================================================================
-constexpr int kFusedThreads = 256, kFusedChunks = 2;
+constexpr int kFusedThreads = 288, kFusedCompute = 256, kFusedIssuer = 256, kFusedChunks = 2;
 constexpr int kFusedSplit = 4, kFusedTilesPerCta = 16;    // a cluster with many pair tiles is shared by up to 4 CTAs
 
 struct FusedSmem {
   static constexpr int D = 128;
-  static constexpr int q = 0, dO = q + kBM * D * 2, k = dO + kBM * D * 2, v = k + kFusedChunks * kBN * D * 2,
-                       p = v + kFusedChunks * kBN * D * 2, g = p + kBM * kBN * 2, stage = g + kBM * kBN * 2,
-                       total = stage + kBM * D * 2 + 1024;      // stage: bf16 dQ rows on their way out
+  static constexpr int kTile = kBM * D * 2;                                // 32 KB
+  static constexpr int q = 0, dO = q + 2 * kTile, k = dO + 2 * kTile, v = k + kFusedChunks * kBN * D * 2,
+                       p = v + kFusedChunks * kBN * D * 2, g = p + kBM * kBN * 2,
+                       total = g + kBM * kBN * 2;   // 224 KB: no slack, the kernel checks the 1024-byte alignment of its base
+  static constexpr int stage = p;                                          // bf16 dQ rows on their way out: the P and G tiles together
   static constexpr uint32_t cS = 0, cDP = 64, cDQ = 128, cDV = 256, cDK = 384, cols = 512;
 };
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* src, bool valid) {
+  const int n = valid ? 16 : 0;                                            // 0 source bytes: the 16 bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(tc::smem_u32(smem_dst)), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
 __global__ void __launch_bounds__(kFusedThreads, 1)
 k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO, const bf16* __restrict__ Kp,
@@ -733,7 +745,10 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   __shared__ uint64_t bar[2];
   __shared__ uint32_t tbase_s;
   __shared__ int32_t pid_s[3][kBM];                        // pair ids of the previous, the current and the next tile
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = tid & 127, wg = tid >> 7;
+  __shared__ int32_t tok_s[2][kBM];                        // tokens of the tile being gathered (alternating slots)
+  __shared__ int err_s;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = tid & 127, wg = (tid >> 7) & 1;
+  const bool cw = warp < 8;                                // compute warp
   const int j = blockIdx.x, sub = blockIdx.y, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
@@ -742,15 +757,26 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   const int k0 = ok[0], kall = ok[dm.SB];
   int ntiles_all = 0;
   for (int pl = 0; pl < dm.SB; ++pl) ntiles_all += (go[(size_t)pl * dm.Ck + 1] - go[(size_t)pl * dm.Ck] + kBM - 1) / kBM;
-  // the tiles of the cluster are dealt round-robin to nsub CTAs (one for all but the most retrieved clusters);
-  // CTAs that share a cluster add their dK, dV with atomics
+  // the tiles of the cluster are dealt round-robin to nsub CTAs (one for all but the most retrieved clusters)
   const int nsub = min(kFusedSplit, max(1, ntiles_all / kFusedTilesPerCta));
   if (ntiles_all == 0 || sub >= nsub) return;
+  if (tc::smem_u32(sm_raw) & 1023u) {                      // the tiles fill the whole dynamic allocation: no room to realign
+    if (tid == 0) atomicExch(status, 2);
+    return;
+  }
+  if (tid == 0) err_s = 0;
   BwdCtx c;
   bwd_setup(c, sm_raw, bar, &tbase_s, SM::cols, tid);
   const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
   const bf16* Kb = Kp + (size_t)pk * dm.N * D; const bf16* Vb = Vp + (size_t)pk * dm.N * D;
   const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
+  // a wait that ran out on one thread ends the walk for all of them at the next barrier
+  auto sync_all = [&]() {
+    if (!c.ok) err_s = 1;
+    tc::fence_before_sync();
+    __syncthreads();
+    if (err_s) c.ok = false;
+  };
   const uint32_t qa = tc::smem_u32(c.sm + SM::q), da = tc::smem_u32(c.sm + SM::dO), ka = tc::smem_u32(c.sm + SM::k),
                  va = tc::smem_u32(c.sm + SM::v), pa = tc::smem_u32(c.sm + SM::p), ga = tc::smem_u32(c.sm + SM::g);
   const uint32_t tl = c.tbase + ((uint32_t)((warp & 3) * 32) << 16);
@@ -778,42 +804,69 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
     };
     auto skip = [&](Item a, int n) { for (int k = 0; k < n; ++k) a = next1(a); return a; };
     auto next_of = [&](const Item& a) { return skip(a, nsub); };         // this CTA's next tile
+    auto chunks_of = [&](const Item& a) {                                 // key chunks of this sweep that the tile's plane sees
+      return a.pl < dm.SB ? (min(KC, max(0, ok[a.pl + 1] - kc0)) + kBN - 1) / kBN : 0;
+    };
     // key / value chunks of this sweep
     __syncthreads();
     const int nkc = min(KC, kall - kc0);                    // keys of the sweep that any plane sees
+    if (cw) {
 #pragma unroll
-    for (int ch = 0; ch < kFusedChunks; ++ch) {
-      const int n = min(kBN, max(0, nkc - ch * kBN));
-      fill_tile<D, kBN, kFusedThreads>(c.sm + SM::k + ch * kBN * D * 2, n, [&](int r) { return Kb + (size_t)(kc0 + ch * kBN + r) * D; }, tid);
-      fill_tile<D, kBN, kFusedThreads>(c.sm + SM::v + ch * kBN * D * 2, n, [&](int r) { return Vb + (size_t)(kc0 + ch * kBN + r) * D; }, tid);
+      for (int ch = 0; ch < kFusedChunks; ++ch) {
+        const int n = min(kBN, max(0, nkc - ch * kBN));
+        fill_tile<D, kBN, kFusedCompute>(c.sm + SM::k + ch * kBN * D * 2, n, [&](int r) { return Kb + (size_t)(kc0 + ch * kBN + r) * D; }, tid);
+        fill_tile<D, kBN, kFusedCompute>(c.sm + SM::v + ch * kBN * D * 2, n, [&](int r) { return Vb + (size_t)(kc0 + ch * kBN + r) * D; }, tid);
+      }
     }
     bool started[kFusedChunks] = {false, false};            // dV^T / dK^T of chunk ch hold something
 
-    TileRegs<D, kBM, kFusedThreads> qreg, oreg;
     float Lreg = 0.f, dreg = 0.f;
-    int pidreg = 0;
+    int pidreg = 0, tokreg = 0;
     auto load_pids = [&](const Item& it) {
-      if (tid < kBM) pidreg = (it.pl < dm.SB && it.t0 + tid < it.g1) ? __ldg(pr + it.t0 + tid) : 0;
+      if (tid < kBM) {
+        pidreg = (it.pl < dm.SB && it.t0 + tid < it.g1) ? __ldg(pr + it.t0 + tid) : 0;
+        tokreg = pidreg / dm.m;
+      }
     };
-    auto load_rows = [&](const Item& it, const int32_t* pid) {
+    // rows of tile `it` (tokens tok[]) into half `b` of the double buffer: thread = 16-byte chunk tid % 16 of
+    // rows tid / 16 + 16 k, so that a warp copies two whole rows per instruction; rows past the end are zeros
+    auto gather_rows = [&](const Item& it, const int32_t* tok, int b) {
       const int nq = min(kBM, it.g1 - it.t0);
-      tile_ldg<D, kBM, kFusedThreads>(qreg, nq, [&](int r) { return Qb + (size_t)(pid[r] / dm.m) * D; }, tid);
-      tile_ldg<D, kBM, kFusedThreads>(oreg, nq, [&](int r) { return dOb + (size_t)(pid[r] / dm.m) * D; }, tid);
-      const size_t tt = (size_t)pq * dm.N + pid[row] / dm.m;
+      const int ck = tid & 15;
+      unsigned char* qd = c.sm + SM::q + b * SM::kTile + (ck >> 3) * kBM * 128;
+      unsigned char* od = c.sm + SM::dO + b * SM::kTile + (ck >> 3) * kBM * 128;
+#pragma unroll
+      for (int k = 0; k < kBM / 16; ++k) {
+        const int r = (tid >> 4) + 16 * k;
+        const size_t at = (size_t)tok[r] * D + ck * 8;
+        cp_async16(qd + tc::sw128_off(r, ck & 7), Qb + at, r < nq);
+        cp_async16(od + tc::sw128_off(r, ck & 7), dOb + at, r < nq);
+      }
+      cp_async_commit();
+      const size_t tt = (size_t)pq * dm.N + tok[row];
       Lreg = row < nq ? LSE[tt] * kLog2e : 0.f;
       dreg = row < nq ? delta[tt] : 0.f;
     };
+    auto issue_first = [&](int b, int ch) {                                // issuer: S = Q K^T and dP = dO V^T for key chunk ch
+      const uint32_t kac = ka + ch * kBN * D * 2, vac = va + ch * kBN * D * 2, qab = qa + b * SM::kTile, dab = da + b * SM::kTile;
+      const uint32_t idesc = tc::idesc_bf16(kBM, kBN, 0, 0);
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase + SM::cS, desc_k<kBM>(qab, ks), desc_k<kBN>(kac, ks), idesc, ks > 0);
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase + SM::cDP, desc_k<kBM>(dab, ks), desc_k<kBN>(vac, ks), idesc, ks > 0);
+      tc::mma_commit(&c.bar[0]);
+    };
     Item cur = skip(first_from(0), sub), nxt = next_of(cur), nn = next_of(nxt);
     load_pids(cur);
-    if (tid < kBM) pid_s[0][tid] = pidreg;
+    if (tid < kBM) { pid_s[0][tid] = pidreg; tok_s[0][tid] = tokreg; }
     load_pids(nxt);
-    __syncthreads();
-    if (cur.pl < dm.SB) load_rows(cur, pid_s[0]);
-    int buf = 0;
+    sync_all();
+    int buf = 0, qb = 0;                                     // slot of the pair-id ring / half of the row double buffer
+    if (cw && cur.pl < dm.SB) gather_rows(cur, tok_s[0], 0);
     // The dQ rows of a tile are written while the first products of the NEXT tile run on the tensor cores
     // (the accumulator columns are only overwritten by that tile's second batch of MMAs).
-    int prev_pid = 0, prev_nq = 0, prev_nch = -1, prev_buf = 0;  // prev_nch < 0: nothing pending
-    auto store_dq = [&]() {
+    int prev_nq = 0, prev_nch = -1, prev_buf = 0;          // prev_nch < 0: nothing pending
+    auto store_dq = [&]() {                                 // compute warps only
       if (prev_nch < 0) return;                                         // uniform over the CTA
       const uint32_t tq = tl + SM::cDQ + wg * (D / 2);
       bf16* base = dq_part + (size_t)pq * dm.N * dm.m * D;
@@ -830,14 +883,14 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
           uint32_t w[4];
 #pragma unroll
           for (int e = 0; e < 4; ++e) {
-            __nv_bfloat162 b2 = prev_nch > 0 ? __floats2bfloat162_rn(v[i + 2 * e] * dm.sigma, v[i + 2 * e + 1] * dm.sigma) : __floats2bfloat162_rn(0.f, 0.f);
+            __nv_bfloat162 b2 = prev_nch > 0 ? __floats2bfloat162_rn(v[i + 2 * e], v[i + 2 * e + 1]) : __floats2bfloat162_rn(0.f, 0.f);
             w[e] = *reinterpret_cast<uint32_t*>(&b2);
           }
           const int ck = (wg * (D / 2) + d0 + i) >> 3;
           *reinterpret_cast<uint4*>(stg + row * 256 + ((ck ^ (row & 15)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
-      __syncthreads();
+      tc::named_bar_sync(1, kFusedCompute);
       if (c.ok) {
 #pragma unroll
         for (int k = 0; k < kBM / 16; ++k) {                            // 8 warps x 8 steps x 2 rows
@@ -856,59 +909,36 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
           }
         }
       }
+      tc::named_bar_sync(1, kFusedCompute);                             // the staging space is the P / G tiles
       prev_nch = -1;
     };
+    bool pre = false;                                       // the first products of the current tile are already issued
     while (cur.pl < dm.SB && c.ok) {
-#ifdef MUSE_PHASE_CLOCKS
-      long long z_ = clock64();
-#define ZCLK(k) { long long n_ = clock64(); c.pc[k] += n_ - z_; z_ = n_; }
-#else
-#define ZCLK(k)
-#endif
       const int nq = min(kBM, cur.g1 - cur.t0);
       const int vis = min(KC, max(0, ok[cur.pl + 1] - kc0));            // keys of this sweep that the plane sees
       const int nch = (vis + kBN - 1) / kBN;
       const int nbuf = buf == 2 ? 0 : buf + 1;
-      tile_sts<D, kBM, kFusedThreads>(qreg, c.sm + SM::q, tid);
-      tile_sts<D, kBM, kFusedThreads>(oreg, c.sm + SM::dO, tid);
-      if (tid < kBM) pid_s[nbuf][tid] = pidreg;                         // pair ids of the next tile
+      const bool pre_next = nch > 0 && chunks_of(nxt) > 0;              // this tile's last barrier also starts the next tile
+      if (tid < kBM) { pid_s[nbuf][tid] = pidreg; tok_s[qb ^ 1][tid] = tokreg; }   // ids of the next tile
       const float L2 = Lreg, dl = dreg;
-      const int my_pid = pid_s[buf][row];
-      tc::fence_async_smem();
-      tc::fence_before_sync();
-      __syncthreads();                                                  // tiles and pid_s[nbuf] visible
-      ZCLK(0)
-      bool prefetched = false;
-      auto prefetch = [&]() {                                           // gathers of the next tile, pair ids of the one after
-        if (prefetched) return;
-        if (nxt.pl < dm.SB) load_rows(nxt, pid_s[nbuf]);
+      if (!pre) {
+        // first tile of the sweep, or the tile before had no key chunk: wait for this tile's rows here
+        if (cw) { cp_async_wait_all(); tc::fence_async_smem(); }
+        sync_all();
+        if (tid == kFusedIssuer && nch > 0 && c.ok) { tc::fence_after_sync(); issue_first(qb, 0); }
+      } else if (cw) {
+        tc::named_bar_sync(1, kFusedCompute);                           // ids of the next tile visible
+      }
+      if (cw) {
+        if (nxt.pl < dm.SB) gather_rows(nxt, tok_s[qb ^ 1], qb ^ 1);      // the other half was last read by the previous tile's MMAs (waited)
         load_pids(nn);
-        prefetched = true;
-      };
-      auto issue_first = [&](int ch) {                                  // S = Q K^T and dP = dO V^T for key chunk ch
-        const uint32_t kac = ka + ch * kBN * D * 2, vac = va + ch * kBN * D * 2;
-        if (tid == 0) {
-          tc::fence_after_sync();
-          const uint32_t idesc = tc::idesc_bf16(kBM, kBN, 0, 0);
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase + SM::cS, desc_k<kBM>(qa, ks), desc_k<kBN>(kac, ks), idesc, ks > 0);
-#pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase + SM::cDP, desc_k<kBM>(da, ks), desc_k<kBN>(vac, ks), idesc, ks > 0);
-          tc::mma_commit(&c.bar[0]);
-        }
-        __syncwarp();
-      };
-      if (nch > 0) issue_first(0);
-      store_dq();                                                       // previous tile's rows leave meanwhile
+        store_dq();                                                     // previous tile's rows leave while the first products run
+      }
       for (int ch = 0; ch < nch && c.ok; ++ch) {
-        const uint32_t kac = ka + ch * kBN * D * 2;
-        if (ch > 0) issue_first(ch);
-        ZCLK(1)
-        if (!tc::mbar_wait(&c.bar[0], c.ph0)) { c.ok = false; break; }
-        c.ph0 ^= 1;
-        tc::fence_after_sync();
-        ZCLK(2)
-        {
+        const bool last = ch + 1 == nch;
+        if (cw) {
+          if (!tc::mbar_wait(&c.bar[0], c.ph0)) c.ok = false;
+          tc::fence_after_sync();
           const int visc = min(kBN, vis - ch * kBN);
           float sv[32], dp[32], pv[32], gv[32];
           tc::tmem_ld32(tl + SM::cS + 32 * wg, sv);
@@ -917,17 +947,22 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
           for (int i = 0; i < 32; ++i) {
             const float e = tc::fast_exp2(sv[i] * scale2 - L2);
             pv[i] = (row < nq && 32 * wg + i < visc) ? e : 0.f;
-            gv[i] = pv[i] * (dp[i] - dl);
+            gv[i] = pv[i] * (dp[i] - dl) * dm.sigma;                    // (sigma rides on G: dQ and dK come out scaled)
+          }
+          if (ch > 0) {                                                 // the previous chunk's MMAs have read P / G
+            if (!tc::mbar_wait(&c.bar[1], c.ph1)) c.ok = false;
+            c.ph1 ^= 1;
           }
           store_row32(c.sm + SM::p, row, wg, pv);
           store_row32(c.sm + SM::g, row, wg, gv);
+          if (last && pre_next) cp_async_wait_all();                    // the next tile's rows, for the products issued below
+          tc::fence_async_smem();
         }
-        ZCLK(3)
-        tc::fence_async_smem();
-        tc::fence_before_sync();
-        __syncthreads();
-        if (tid == 0) {
+        c.ph0 ^= 1;
+        sync_all();
+        if (tid == kFusedIssuer && c.ok) {
           tc::fence_after_sync();
+          const uint32_t kac = ka + ch * kBN * D * 2, qab = qa + qb * SM::kTile, dab = da + qb * SM::kTile;
           const uint32_t id_dq = tc::idesc_bf16(kBM, D, 0, 1);          // A = G (contraction over keys), B = key rows MN-major
           const uint32_t id_t = tc::idesc_bf16(D, kBN, 1, 1);           // A = dO / Q tile and B = P / G tile, both contracted over pairs
 #pragma unroll
@@ -935,61 +970,51 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
             tc::mma_bf16_ss(c.tbase + SM::cDQ, tc::smem_desc_sw128(ga + ks * 32, 16, 1024), desc_mn<kBN>(kac, ks), id_dq, ch > 0 || ks > 0);
 #pragma unroll
           for (int ks = 0; ks < kBM / 16; ++ks)
-            tc::mma_bf16_ss(c.tbase + SM::cDV + ch * kBN, desc_mn<kBM>(da, ks), tc::smem_desc_sw128(pa + ks * 16 * 128, kBM * 128, 1024), id_t,
+            tc::mma_bf16_ss(c.tbase + SM::cDV + ch * kBN, desc_mn<kBM>(dab, ks), tc::smem_desc_sw128(pa + ks * 16 * 128, kBM * 128, 1024), id_t,
                             started[ch] || ks > 0);
 #pragma unroll
           for (int ks = 0; ks < kBM / 16; ++ks)
-            tc::mma_bf16_ss(c.tbase + SM::cDK + ch * kBN, desc_mn<kBM>(qa, ks), tc::smem_desc_sw128(ga + ks * 16 * 128, kBM * 128, 1024), id_t,
+            tc::mma_bf16_ss(c.tbase + SM::cDK + ch * kBN, desc_mn<kBM>(qab, ks), tc::smem_desc_sw128(ga + ks * 16 * 128, kBM * 128, 1024), id_t,
                             started[ch] || ks > 0);
           tc::mma_commit(&c.bar[1]);
+          // queued behind them: the first products of the next chunk, or of the next tile
+          if (!last) issue_first(qb, ch + 1);
+          else if (pre_next) issue_first(qb ^ 1, 0);
         }
         started[ch] = true;
-        __syncwarp();
-        prefetch();                                                     // the gathers are issued while these MMAs run
-        ZCLK(4)
-        if (!tc::mbar_wait(&c.bar[1], c.ph1)) { c.ok = false; break; }
+      }
+      if (cw && nch > 0) {                                              // the last chunk's MMAs: dQ complete, both halves of the buffers free
+        if (!tc::mbar_wait(&c.bar[1], c.ph1)) c.ok = false;
         c.ph1 ^= 1;
         tc::fence_after_sync();
-        ZCLK(5)
       }
-      prefetch();
-      prev_pid = my_pid; prev_nq = nq; prev_nch = nch; prev_buf = buf;
+      pre = pre_next;
+      prev_nq = nq; prev_nch = nch; prev_buf = buf;
       tc::fence_before_sync();
-      cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf;
-      ZCLK(6)
-#ifdef MUSE_PHASE_CLOCKS
-      c.pc[7] += 1;
-#endif
+      cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf; qb ^= 1;
     }
-    store_dq();
-    // dV (warpgroup 0) and dK (warpgroup 1) of this sweep's keys: thread = output dim, one key per column
+    if (cw) {
+      store_dq();
+      // dV (warpgroup 0) and dK (warpgroup 1) of this sweep's keys: thread = output dim, one key per column
 #pragma unroll
-    for (int ch = 0; ch < kFusedChunks; ++ch) {
-      if (!started[ch]) continue;                                       // uniform over the CTA
-      const int n = min(kBN, nkc - ch * kBN);
-      float* dst = (wg == 0 ? dV_perm : dK_perm) + ((size_t)pq * dm.N + kc0 + ch * kBN) * D + row;
-      const float f = wg == 0 ? 1.f : dm.sigma;
+      for (int ch = 0; ch < kFusedChunks; ++ch) {
+        if (!started[ch]) continue;                                     // uniform over the CTA
+        const int n = min(kBN, nkc - ch * kBN);
+        float* dst = (wg == 0 ? dV_perm : dK_perm) + ((size_t)pq * dm.N + kc0 + ch * kBN) * D + row;
 #pragma unroll
-      for (int u0 = 0; u0 < kBN; u0 += 32) {
-        float v[32];
-        tc::tmem_ld32(tl + (wg == 0 ? SM::cDV : SM::cDK) + ch * kBN + u0, v);
-        if (c.ok) {
+        for (int u0 = 0; u0 < kBN; u0 += 32) {
+          float v[32];
+          tc::tmem_ld32(tl + (wg == 0 ? SM::cDV : SM::cDK) + ch * kBN + u0, v);
+          if (c.ok) {
 #pragma unroll
-          for (int u = 0; u < 32; ++u) {
-            if (u0 + u < n) {
-              if (nsub > 1) atomicAdd(dst + (size_t)(u0 + u) * D, v[u] * f);
-              else dst[(size_t)(u0 + u) * D] += v[u] * f;
-            }
+            for (int u = 0; u < 32; ++u)
+              if (u0 + u < n) atomicAdd(dst + (size_t)(u0 + u) * D, v[u]);       // (result unused: no round trip)
           }
         }
       }
     }
     tc::fence_before_sync();
   }
-#ifdef MUSE_PHASE_CLOCKS
-  if (tid == 0 && c.pc[7] >= 12 && atomicCAS(status + 40, 0, 1) == 0)
-    for (int k = 0; k < 8; ++k) status[41 + k] = (int)c.pc[k];
-#endif
   bwd_teardown(c, SM::cols, tid, status);
 }
 
