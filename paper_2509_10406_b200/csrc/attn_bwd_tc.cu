@@ -708,13 +708,15 @@ k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
 //   dQ   += G K                     [pairs][D]   written per pair as a bf16 row
 //   dV^T += dO^T P,  dK^T += Q^T G  [D][keys]    accumulated in TMEM over all tiles and planes
 // Eight warps do the arithmetic; lane 0 of a ninth warp issues every MMA, so that the first
-// products of the next chunk (or tile) queue behind the second batch of the current one.  The Q and
-// dO rows of a tile are gathered once for all three products, one tile ahead, by asynchronous
-// 16-byte copies straight into the other half of a double buffer; pair ids run two tiles ahead,
-// across plane boundaries.  The CTA owns the cluster's keys for its head (or shares them with up
+// products of the next chunk (or tile) queue behind the second batch of the current one; three
+// more warps gather.  The Q and dO rows of a tile are gathered once for all three products, one
+// tile ahead, by asynchronous 16-byte copies straight into the other half of a double buffer (the
+// load/store unit takes a few thousand cycles to accept a tile's 4096 copies: time the arithmetic
+// warps do not have); pair ids run two tiles ahead, across plane boundaries.  The CTA owns the cluster's keys for its head (or shares them with up
 // to three others): dK and dV leave as fire-and-forget adds, thread = output dim.
 // ================================================================================================
-constexpr int kFusedThreads = 288, kFusedCompute = 256, kFusedIssuer = 256, kFusedChunks = 2;
+constexpr int kFusedThreads = 384, kFusedCompute = 256, kFusedIssuer = 256, kFusedChunks = 2;
+constexpr int kFusedGather0 = 288, kFusedGather = 96;    // warps 9-11 gather rows; warps 0-8 meet at barrier 2, warps 0-7 and 9-11 at barrier 1
 constexpr int kFusedSplit = 4, kFusedTilesPerCta = 16;    // a cluster with many pair tiles is shared by up to 4 CTAs
 
 struct FusedSmem {
@@ -742,13 +744,13 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   typedef FusedSmem SM;
   constexpr int D = SM::D, KC = kFusedChunks * kBN;        // keys per sweep
   extern __shared__ __align__(1024) unsigned char sm_raw[];
-  __shared__ uint64_t bar[2];
+  __shared__ uint64_t bar[2], bar_rows[2];                 // bar_rows[b]: half b of the row double buffer is filled
   __shared__ uint32_t tbase_s;
   __shared__ int32_t pid_s[3][kBM];                        // pair ids of the previous, the current and the next tile
   __shared__ int32_t tok_s[2][kBM];                        // tokens of the tile being gathered (alternating slots)
   __shared__ int err_s;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = tid & 127, wg = (tid >> 7) & 1;
-  const bool cw = warp < 8;                                // compute warp
+  const bool cw = warp < 8, gw = warp >= 9;                // compute warp / gather warp
   const int j = blockIdx.x, sub = blockIdx.y, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
@@ -764,18 +766,25 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
     if (tid == 0) atomicExch(status, 2);
     return;
   }
-  if (tid == 0) err_s = 0;
+  if (tid == 0) { err_s = 0; tc::mbar_init(&bar_rows[0], kFusedGather); tc::mbar_init(&bar_rows[1], kFusedGather); }
+  uint32_t ph_rows[2] = {0, 0};
   BwdCtx c;
   bwd_setup(c, sm_raw, bar, &tbase_s, SM::cols, tid);
   const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
   const bf16* Kb = Kp + (size_t)pk * dm.N * D; const bf16* Vb = Vp + (size_t)pk * dm.N * D;
   const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
   // a wait that ran out on one thread ends the walk for all of them at the next barrier
-  auto sync_all = [&]() {
+  auto sync_all = [&]() {                                  // arithmetic warps and the issuing warp
     if (!c.ok) err_s = 1;
     tc::fence_before_sync();
-    __syncthreads();
+    tc::named_bar_sync(2, kFusedCompute + 32);
     if (err_s) c.ok = false;
+  };
+  // Every warp walks the same sequence of tiles to the end, whatever happens (after a wait ran out the
+  // remaining waits are skipped): the barriers below always see all their warps.
+  auto wait_rows = [&](int b) {
+    if (c.ok && !tc::mbar_wait(&bar_rows[b], ph_rows[b])) c.ok = false;
+    ph_rows[b] ^= 1;
   };
   const uint32_t qa = tc::smem_u32(c.sm + SM::q), da = tc::smem_u32(c.sm + SM::dO), ka = tc::smem_u32(c.sm + SM::k),
                  va = tc::smem_u32(c.sm + SM::v), pa = tc::smem_u32(c.sm + SM::p), ga = tc::smem_u32(c.sm + SM::g);
@@ -785,7 +794,7 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   // work items: (plane, first pair of the tile); a plane takes part in a sweep if it has pairs and, from the
   // second sweep on, if it sees keys of that sweep
   struct Item { int pl, t0, g1; };
-  for (int kc0 = k0; (kc0 < kall || kc0 == k0) && c.ok; kc0 += KC) {
+  for (int kc0 = k0; kc0 < kall || kc0 == k0; kc0 += KC) {
     const bool first_sweep = kc0 == k0;
     auto plane_active = [&](int pl) {
       const int g0 = go[(size_t)pl * dm.Ck], g1 = go[(size_t)pl * dm.Ck + 1];
@@ -828,21 +837,27 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
         tokreg = pidreg / dm.m;
       }
     };
-    // rows of tile `it` (tokens tok[]) into half `b` of the double buffer: thread = 16-byte chunk tid % 16 of
-    // rows tid / 16 + 16 k, so that a warp copies two whole rows per instruction; rows past the end are zeros
+    // gather warps: rows of tile `it` (tokens tok[]) into half `b` of the double buffer; thread = 16-byte chunk
+    // g % 16 of rows g / 16 + 6 k, so that a warp copies two whole rows per instruction; rows past the end are zeros
     auto gather_rows = [&](const Item& it, const int32_t* tok, int b) {
       const int nq = min(kBM, it.g1 - it.t0);
-      const int ck = tid & 15;
+      const int g = tid - kFusedGather0, ck = g & 15;
       unsigned char* qd = c.sm + SM::q + b * SM::kTile + (ck >> 3) * kBM * 128;
       unsigned char* od = c.sm + SM::dO + b * SM::kTile + (ck >> 3) * kBM * 128;
-#pragma unroll
-      for (int k = 0; k < kBM / 16; ++k) {
-        const int r = (tid >> 4) + 16 * k;
+#pragma unroll 2
+      for (int r = g >> 4; r < kBM; r += kFusedGather / 16) {
         const size_t at = (size_t)tok[r] * D + ck * 8;
         cp_async16(qd + tc::sw128_off(r, ck & 7), Qb + at, r < nq);
         cp_async16(od + tc::sw128_off(r, ck & 7), dOb + at, r < nq);
       }
       cp_async_commit();
+      cp_async_wait_all();
+      tc::fence_async_smem();                               // the tensor cores read the rows through the async proxy
+      tc::mbar_arrive(&bar_rows[b]);
+    };
+    // arithmetic warps: L and delta of the tile's rows, one tile ahead
+    auto load_row_scalars = [&](const Item& it, const int32_t* tok) {
+      const int nq = min(kBM, it.g1 - it.t0);
       const size_t tt = (size_t)pq * dm.N + tok[row];
       Lreg = row < nq ? LSE[tt] * kLog2e : 0.f;
       dreg = row < nq ? delta[tt] : 0.f;
@@ -860,9 +875,12 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
     load_pids(cur);
     if (tid < kBM) { pid_s[0][tid] = pidreg; tok_s[0][tid] = tokreg; }
     load_pids(nxt);
-    sync_all();
+    __syncthreads();
     int buf = 0, qb = 0;                                     // slot of the pair-id ring / half of the row double buffer
-    if (cw && cur.pl < dm.SB) gather_rows(cur, tok_s[0], 0);
+    if (cur.pl < dm.SB) {
+      if (gw) gather_rows(cur, tok_s[0], 0);
+      if (cw) load_row_scalars(cur, tok_s[0]);
+    }
     // The dQ rows of a tile are written while the first products of the NEXT tile run on the tensor cores
     // (the accumulator columns are only overwritten by that tile's second batch of MMAs).
     int prev_nq = 0, prev_nch = -1, prev_buf = 0;          // prev_nch < 0: nothing pending
@@ -890,7 +908,7 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
           *reinterpret_cast<uint4*>(stg + row * 256 + ((ck ^ (row & 15)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
       }
-      tc::named_bar_sync(1, kFusedCompute);
+      tc::named_bar_sync(3, kFusedCompute);
       if (c.ok) {
 #pragma unroll
         for (int k = 0; k < kBM / 16; ++k) {                            // 8 warps x 8 steps x 2 rows
@@ -909,11 +927,17 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
           }
         }
       }
-      tc::named_bar_sync(1, kFusedCompute);                             // the staging space is the P / G tiles
+      tc::named_bar_sync(3, kFusedCompute);                             // the staging space is the P / G tiles
       prev_nch = -1;
     };
     bool pre = false;                                       // the first products of the current tile are already issued
-    while (cur.pl < dm.SB && c.ok) {
+    while (cur.pl < dm.SB) {
+#ifdef MUSE_PHASE_CLOCKS
+      long long z_ = clock64();
+#define ZCLK(k) { long long n_ = clock64(); c.pc[k] += n_ - z_; z_ = n_; }
+#else
+#define ZCLK(k)
+#endif
       const int nq = min(kBM, cur.g1 - cur.t0);
       const int vis = min(KC, max(0, ok[cur.pl + 1] - kc0));            // keys of this sweep that the plane sees
       const int nch = (vis + kBN - 1) / kBN;
@@ -921,24 +945,33 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       const bool pre_next = nch > 0 && chunks_of(nxt) > 0;              // this tile's last barrier also starts the next tile
       if (tid < kBM) { pid_s[nbuf][tid] = pidreg; tok_s[qb ^ 1][tid] = tokreg; }   // ids of the next tile
       const float L2 = Lreg, dl = dreg;
+      // ids of the next tile visible to the gather warps; the other half of the row buffer was last read by the
+      // previous tile's MMAs, which the arithmetic warps have waited for
+      if (cw || gw) tc::named_bar_sync(1, kFusedCompute + kFusedGather);
+      if (gw) {
+        if (nxt.pl < dm.SB) gather_rows(nxt, tok_s[qb ^ 1], qb ^ 1);
+        cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf; qb ^= 1;
+        continue;
+      }
       if (!pre) {
         // first tile of the sweep, or the tile before had no key chunk: wait for this tile's rows here
-        if (cw) { cp_async_wait_all(); tc::fence_async_smem(); }
+        if (cw) { wait_rows(qb); tc::fence_async_smem(); }
         sync_all();
-        if (tid == kFusedIssuer && nch > 0 && c.ok) { tc::fence_after_sync(); issue_first(qb, 0); }
-      } else if (cw) {
-        tc::named_bar_sync(1, kFusedCompute);                           // ids of the next tile visible
+        if (tid == kFusedIssuer && nch > 0) { tc::fence_after_sync(); issue_first(qb, 0); }
       }
+      ZCLK(0)
       if (cw) {
-        if (nxt.pl < dm.SB) gather_rows(nxt, tok_s[qb ^ 1], qb ^ 1);      // the other half was last read by the previous tile's MMAs (waited)
+        if (nxt.pl < dm.SB) load_row_scalars(nxt, tok_s[qb ^ 1]);
         load_pids(nn);
         store_dq();                                                     // previous tile's rows leave while the first products run
       }
-      for (int ch = 0; ch < nch && c.ok; ++ch) {
+      ZCLK(1)
+      for (int ch = 0; ch < nch; ++ch) {
         const bool last = ch + 1 == nch;
         if (cw) {
-          if (!tc::mbar_wait(&c.bar[0], c.ph0)) c.ok = false;
+          if (c.ok && !tc::mbar_wait(&c.bar[0], c.ph0)) c.ok = false;
           tc::fence_after_sync();
+          ZCLK(2)
           const int visc = min(kBN, vis - ch * kBN);
           float sv[32], dp[32], pv[32], gv[32];
           tc::tmem_ld32(tl + SM::cS + 32 * wg, sv);
@@ -950,17 +983,20 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
             gv[i] = pv[i] * (dp[i] - dl) * dm.sigma;                    // (sigma rides on G: dQ and dK come out scaled)
           }
           if (ch > 0) {                                                 // the previous chunk's MMAs have read P / G
-            if (!tc::mbar_wait(&c.bar[1], c.ph1)) c.ok = false;
+            if (c.ok && !tc::mbar_wait(&c.bar[1], c.ph1)) c.ok = false;
             c.ph1 ^= 1;
           }
           store_row32(c.sm + SM::p, row, wg, pv);
           store_row32(c.sm + SM::g, row, wg, gv);
-          if (last && pre_next) cp_async_wait_all();                    // the next tile's rows, for the products issued below
+          ZCLK(3)
+          if (last && pre_next) wait_rows(qb ^ 1);                      // the next tile's rows, for the products issued below
           tc::fence_async_smem();
+          ZCLK(4)
         }
         c.ph0 ^= 1;
         sync_all();
-        if (tid == kFusedIssuer && c.ok) {
+        ZCLK(5)
+        if (tid == kFusedIssuer) {
           tc::fence_after_sync();
           const uint32_t kac = ka + ch * kBN * D * 2, qab = qa + qb * SM::kTile, dab = da + qb * SM::kTile;
           const uint32_t id_dq = tc::idesc_bf16(kBM, D, 0, 1);          // A = G (contraction over keys), B = key rows MN-major
@@ -984,10 +1020,14 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
         started[ch] = true;
       }
       if (cw && nch > 0) {                                              // the last chunk's MMAs: dQ complete, both halves of the buffers free
-        if (!tc::mbar_wait(&c.bar[1], c.ph1)) c.ok = false;
+        if (c.ok && !tc::mbar_wait(&c.bar[1], c.ph1)) c.ok = false;
         c.ph1 ^= 1;
         tc::fence_after_sync();
       }
+      ZCLK(5)
+#ifdef MUSE_PHASE_CLOCKS
+      c.pc[7] += 1;
+#endif
       pre = pre_next;
       prev_nq = nq; prev_nch = nch; prev_buf = buf;
       tc::fence_before_sync();
@@ -1015,6 +1055,10 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
     }
     tc::fence_before_sync();
   }
+#ifdef MUSE_PHASE_CLOCKS
+  if (tid == 0 && c.pc[7] >= 12 && atomicCAS(status + 40, 0, 1) == 0)
+    for (int k = 0; k < 8; ++k) status[41 + k] = (int)c.pc[k];
+#endif
   bwd_teardown(c, SM::cols, tid, status);
 }
 
