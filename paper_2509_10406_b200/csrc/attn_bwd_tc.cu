@@ -742,6 +742,10 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
                    const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
                    bf16* __restrict__ dq_part, float* __restrict__ dK_perm, float* __restrict__ dV_perm, int* __restrict__ status) {
   typedef FusedSmem SM;
+#ifdef MUSE_PHASE_CLOCKS
+  const long long t_in_ = clock64();
+  long long t_l0_ = 0, t_l1_ = 0, t_pre_ = 0;
+#endif
   constexpr int D = SM::D, KC = kFusedChunks * kBN;        // keys per sweep
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar[2], bar_rows[2];                 // bar_rows[b]: half b of the row double buffer is filled
@@ -770,6 +774,9 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   uint32_t ph_rows[2] = {0, 0};
   BwdCtx c;
   bwd_setup(c, sm_raw, bar, &tbase_s, SM::cols, tid);
+#ifdef MUSE_PHASE_CLOCKS
+  t_pre_ = clock64();
+#endif
   const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
   const bf16* Kb = Kp + (size_t)pk * dm.N * D; const bf16* Vb = Vp + (size_t)pk * dm.N * D;
   const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
@@ -930,6 +937,9 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       tc::named_bar_sync(3, kFusedCompute);                             // the staging space is the P / G tiles
       prev_nch = -1;
     };
+#ifdef MUSE_PHASE_CLOCKS
+    t_l0_ = clock64();
+#endif
     bool pre = false;                                       // the first products of the current tile are already issued
     while (cur.pl < dm.SB) {
 #ifdef MUSE_PHASE_CLOCKS
@@ -1033,6 +1043,9 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       tc::fence_before_sync();
       cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf; qb ^= 1;
     }
+#ifdef MUSE_PHASE_CLOCKS
+    t_l1_ = clock64();
+#endif
     if (cw) {
       store_dq();
       // dV (warpgroup 0) and dK (warpgroup 1) of this sweep's keys: thread = output dim, one key per column
@@ -1057,7 +1070,10 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   }
 #ifdef MUSE_PHASE_CLOCKS
   if (tid == 0 && c.pc[7] >= 12 && atomicCAS(status + 40, 0, 1) == 0)
+  {
     for (int k = 0; k < 8; ++k) status[41 + k] = (int)c.pc[k];
+    status[49] = (int)(t_pre_ - t_in_); status[50] = (int)(t_l0_ - t_in_); status[51] = (int)(t_l1_ - t_l0_); status[52] = (int)(clock64() - t_l1_);
+  }
 #endif
   bwd_teardown(c, SM::cols, tid, status);
 }
