@@ -400,20 +400,28 @@ k_ret_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, c
 // ---- exact retrieval, cluster-resident version (D = 128) ---------------------------------------------
 // One CTA per (key cluster j, head): 128 of the cluster's keys and values stay in shared memory (two
 // chunks of 64) while the CTA walks the retrieving (query, slot) pairs of every plane in tiles of 128.
-// All logits of a tile come from one batch of MMAs, so the softmax needs no running rescale; the Q rows
-// of the next tile are gathered (registers) and the finished rows of the previous tile are written
-// (staged, whole 256-byte rows) while the tensor core works on the current one.  A cluster with more
-// than 128 visible keys takes further sweeps, whose partial results are merged into the stored rows by
-// their log-sum-exp weights.
-constexpr int kRcThreads = 256, kRcKeys = 128;
+// All logits of a tile come from one batch of MMAs, so the softmax needs no running rescale.  Eight
+// warps do the softmax and write the finished rows (staged, whole 256-byte rows); lane 0 of a ninth
+// warp issues every MMA, the logits of the next tile queued right behind the P V product of the
+// current one, whose output alternates between two accumulators so that nobody waits for it; three
+// more warps gather the Q rows one tile ahead, by asynchronous 16-byte copies into the other half of
+// a double buffer.  A cluster with more than 128 visible keys takes further sweeps, whose partial
+// results are merged into the stored rows by their log-sum-exp weights.
+constexpr int kRcThreads = 384, kRcCompute = 256, kRcIssuer = 256, kRcGather0 = 288, kRcGather = 96, kRcKeys = 128;
 constexpr int kRcSplit = 4, kRcTilesPerCta = 16;          // a cluster with many pair tiles is shared by up to 4 CTAs
 
 struct RcSmem {
   static constexpr int D = 128;
-  static constexpr int q = 0, k = q + kTcM * D * 2, v = k + kRcKeys * D * 2, p = v + kRcKeys * D * 2,
-                       stage = p + 2 * kTcM * kTcN * 2, total = stage + kTcM * D * 2 + 1024;
-  static constexpr uint32_t cS = 0, cO = 128, cols = 256;
+  static constexpr int kTile = kTcM * D * 2;               // 32 KB
+  static constexpr int q = 0, k = q + 2 * kTile, v = k + kRcKeys * D * 2, p = v + kRcKeys * D * 2,
+                       stage = p + 2 * kTcM * kTcN * 2, total = stage + kTile + 1024;
+  static constexpr uint32_t cS = 0, cO = 128, cols = 512;  // S (two chunks) | O of even tiles | O of odd tiles
 };
+
+__device__ __forceinline__ void rc_cp_async16(void* smem_dst, const void* src, bool valid) {
+  const int n = valid ? 16 : 0;                            // 0 source bytes: the 16 bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(tc::smem_u32(smem_dst)), "l"(src), "r"(n) : "memory");
+}
 
 __global__ void __launch_bounds__(kRcThreads, 1)
 k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, const bf16* __restrict__ Vp,
@@ -422,11 +430,14 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   typedef RcSmem SM;
   constexpr int D = SM::D;
   extern __shared__ __align__(1024) unsigned char sm_raw[];
-  __shared__ uint64_t bar[2];
+  __shared__ uint64_t bar[2], bar_rows[2];                 // S ready / P V done / half b of the Q double buffer filled
   __shared__ uint32_t tbase_s;
   __shared__ int32_t pid_s[3][kTcM];                       // pair ids of the previous, the current and the next tile
+  __shared__ int32_t tok_s[2][kTcM];                       // tokens of the tile being gathered (alternating slots)
   __shared__ float mx_s[2][kTcM], sum_s[2][kTcM], wold_s[kTcM], wnew_s[kTcM];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = tid & 127, wg = tid >> 7;
+  __shared__ int err_s;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = tid & 127, wg = (tid >> 7) & 1;
+  const bool cw = warp < 8, gw = warp >= 9;                // softmax warp / gather warp
   const int j = blockIdx.x, sub = blockIdx.y, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
@@ -441,7 +452,12 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
 
   unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
   if (warp == 0) tc::tmem_alloc(&tbase_s, SM::cols);
-  if (tid == 0) { tc::mbar_init(&bar[0], 1); tc::mbar_init(&bar[1], 1); tc::mbar_init_fence(); }
+  if (tid == 0) {
+    tc::mbar_init(&bar[0], 1); tc::mbar_init(&bar[1], 1);
+    tc::mbar_init(&bar_rows[0], kRcGather); tc::mbar_init(&bar_rows[1], kRcGather);
+    tc::mbar_init_fence();
+    err_s = 0;
+  }
   const bf16* Qb = Q + (size_t)pq * dm.N * D;
   const bf16* Kb = Kp + (size_t)pk * dm.N * D;
   const bf16* Vb = Vp + (size_t)pk * dm.N * D;
@@ -453,8 +469,20 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   const uint32_t tbase = tbase_s, tl = tbase + ((uint32_t)((warp & 3) * 32) << 16);
   const uint32_t qa = tc::smem_u32(sm + SM::q), ka = tc::smem_u32(sm + SM::k), va = tc::smem_u32(sm + SM::v), pa = tc::smem_u32(sm + SM::p);
   const float scale2 = dm.sigma * 1.4426950408889634f;
-  uint32_t ph0 = 0, ph1 = 0;
+  uint32_t ph0 = 0, ph1 = 0, ph_rows[2] = {0, 0};
   bool ok_ = true;
+  // Every warp walks the same sequence of tiles to the end, whatever happens (after a wait ran out the
+  // remaining waits are skipped), so the barriers below always see all their warps.
+  auto sync_cw_issuer = [&]() {                            // softmax warps and the issuing warp
+    if (!ok_) err_s = 1;
+    tc::fence_before_sync();
+    tc::named_bar_sync(2, kRcCompute + 32);
+    if (err_s) ok_ = false;
+  };
+  auto wait_rows = [&](int b) {
+    if (ok_ && !tc::mbar_wait(&bar_rows[b], ph_rows[b])) ok_ = false;
+    ph_rows[b] ^= 1;
+  };
 
   struct Item { int pl, t0, g1; };
   int kc0 = k0;                                             // first key of the current sweep
@@ -472,30 +500,63 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   };
   auto skip = [&](Item a, int n) { for (int k = 0; k < n; ++k) a = next1(a); return a; };
   auto next_of = [&](const Item& a) { return skip(a, nsub); };           // this CTA's next tile
-  uint4 qreg[kTcM * (D / 8) / kRcThreads];                 // the next tile's Q rows between their loads and their stores
-  int pidreg = 0;
-  auto load_pids = [&](const Item& it) {
-    if (tid < kTcM) pidreg = (it.pl < dm.SB && it.t0 + tid < it.g1) ? __ldg(pr + it.t0 + tid) : 0;
+  auto chunks_of = [&](const Item& a) {                                   // key chunks of this sweep that the tile's plane sees
+    return a.pl < dm.SB ? (min(kRcKeys, max(0, ok[a.pl + 1] - kc0)) + kTcN - 1) / kTcN : 0;
   };
-  auto load_rows = [&](const Item& it, const int32_t* pid) {
-    const int nq = min(kTcM, it.g1 - it.t0);
-#pragma unroll
-    for (int k = 0; k < kTcM * (D / 8) / kRcThreads; ++k) {
-      const int e = tid + kRcThreads * k, r = e / (D / 8), ck = e % (D / 8);
-      qreg[k] = r < nq ? __ldg(reinterpret_cast<const uint4*>(Qb + (size_t)(pid[r] / dm.m) * D) + ck) : make_uint4(0u, 0u, 0u, 0u);
+  int pidreg = 0, tokreg = 0;
+  auto load_pids = [&](const Item& it) {
+    if (tid < kTcM) {
+      pidreg = (it.pl < dm.SB && it.t0 + tid < it.g1) ? __ldg(pr + it.t0 + tid) : 0;
+      tokreg = pidreg / dm.m;
     }
   };
-  // finished rows of the previous tile: normalised, bf16, staged, then stored 16 lanes per row
-  int prev_nq = 0, prev_buf = 0;
+  // gather warps: Q rows of tile `it` (tokens tok[]) into half `b`; thread = 16-byte chunk g % 16 of rows
+  // g / 16 + 6 k, so that a warp copies two whole rows per instruction; rows past the end are zeros
+  auto gather_rows = [&](const Item& it, const int32_t* tok, int b) {
+    const int nq = min(kTcM, it.g1 - it.t0);
+    const int g = tid - kRcGather0, ck = g & 15;
+    unsigned char* qd = sm + SM::q + b * SM::kTile + (ck >> 3) * kTcM * 128;
+#pragma unroll 2
+    for (int r = g >> 4; r < kTcM; r += kRcGather / 16)
+      rc_cp_async16(qd + tc::sw128_off(r, ck & 7), Qb + (size_t)tok[r] * D + ck * 8, r < nq);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    tc::fence_async_smem();                                 // the tensor cores read the rows through the async proxy
+    tc::mbar_arrive(&bar_rows[b]);
+  };
+  auto issue_s = [&](int b, int nch) {                      // issuer: logits of the tile whose rows are in half b
+    const uint32_t idesc = tc::idesc_bf16(kTcM, kTcN, 0, 0);
+    const uint32_t qab = qa + b * SM::kTile;
+    for (int ch = 0; ch < nch; ++ch) {
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks)
+        tc::mma_bf16_ss(tbase + SM::cS + ch * kTcN, tc::smem_desc_sw128(qab + (ks / 4) * kTcM * 128 + (ks % 4) * 32, 16, 1024),
+                        tc::smem_desc_sw128(ka + ch * kTcN * D * 2 + (ks / 4) * kTcN * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
+    }
+    tc::mma_commit(&bar[0]);
+  };
+  // finished rows of the previous tile: normalised, bf16, staged, then stored 16 lanes per row (softmax warps)
+  int prev_nq = 0, prev_buf = 0, prev_o = 0;
   float prev_inv = 0.f, prev_lse = 0.f;
   bool pending = false, prev_first = true;
+  // The P V product of a tile is waited for before the next one can be issued (a parity wait must not fall
+  // two phases behind its barrier): by the next tile's softmax before it overwrites P, or by the deferred store.
+  bool pv_pending = false;
+  auto wait_pv = [&]() {
+    if (!pv_pending) return;                              // uniform over the CTA
+    if (ok_ && !tc::mbar_wait(&bar[1], ph1)) ok_ = false;
+    ph1 ^= 1;
+    tc::fence_after_sync();
+    pv_pending = false;
+  };
   auto store_prev = [&]() {
     if (!pending) return;                                 // uniform over the CTA
     unsigned char* stg = sm + SM::stage;
+    wait_pv();
 #pragma unroll
     for (int d0 = 0; d0 < D / 2; d0 += 32) {
       float v[32];
-      tc::tmem_ld32(tl + SM::cO + wg * (D / 2) + d0, v);
+      tc::tmem_ld32(tl + SM::cO + prev_o * D + wg * (D / 2) + d0, v);
 #pragma unroll
       for (int i = 0; i < 32; i += 8) {
         uint32_t w[4];
@@ -522,7 +583,7 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
         *lp = tot > 0.f ? mxl + __logf(tot) : -INFINITY;
       }
     }
-    __syncthreads();
+    tc::named_bar_sync(3, kRcCompute);
     if (ok_) {
       bf16* base = o_part + (size_t)pq * dm.N * dm.m * D;
 #pragma unroll
@@ -547,133 +608,136 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
     pending = false;
   };
 
-  for (; (kc0 < kall || first_sweep) && ok_; kc0 += kRcKeys, first_sweep = false) {
-  __syncthreads();                                          // the previous sweep is done with the key / value tiles
-  // the cluster's keys (K-major for S = Q K^T) and values (MN-major for O = P V), two chunks of 64
-  for (int ch = 0; ch < 2; ++ch) {
-    const int n = min(kTcN, max(0, kall - kc0 - ch * kTcN));
-    for (int e = tid; e < kTcN * (D / 8); e += kRcThreads) {
-      const int r = e / (D / 8), ck = e % (D / 8);
-      uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
-      if (r < n) {
-        a = reinterpret_cast<const uint4*>(Kb + (size_t)(kc0 + ch * kTcN + r) * D)[ck];
-        b = reinterpret_cast<const uint4*>(Vb + (size_t)(kc0 + ch * kTcN + r) * D)[ck];
-      }
-      const uint32_t off = ch * kTcN * D * 2 + (ck >> 3) * kTcN * 128 + tc::sw128_off(r, ck & 7);
-      *reinterpret_cast<uint4*>(sm + SM::k + off) = a;
-      *reinterpret_cast<uint4*>(sm + SM::v + off) = b;
-    }
-  }
-  tc::fence_async_smem();
-  Item cur = skip(first_from(0), sub), nxt = next_of(cur), nn = next_of(nxt);
-  load_pids(cur);
-  if (tid < kTcM) pid_s[0][tid] = pidreg;
-  load_pids(nxt);
-  __syncthreads();
-  if (cur.pl < dm.SB) load_rows(cur, pid_s[0]);
-  int buf = 0;
-  while (cur.pl < dm.SB && ok_) {
-    const int nq = min(kTcM, cur.g1 - cur.t0);
-    const int vis = min(kRcKeys, max(0, ok[cur.pl + 1] - kc0));   // keys of this sweep that the plane sees
-    const int nch = (vis + kTcN - 1) / kTcN;
-    const int nbuf = buf == 2 ? 0 : buf + 1;
-#pragma unroll
-    for (int k = 0; k < kTcM * (D / 8) / kRcThreads; ++k) {
-      const int e = tid + kRcThreads * k, r = e / (D / 8), ck = e % (D / 8);
-      *reinterpret_cast<uint4*>(sm + SM::q + (ck >> 3) * kTcM * 128 + tc::sw128_off(r, ck & 7)) = qreg[k];
-    }
-    if (tid < kTcM) pid_s[nbuf][tid] = pidreg;              // pair ids of the next tile
-    tc::fence_async_smem();
-    tc::fence_before_sync();
-    __syncthreads();
-    if (tid == 0 && nch > 0) {
-      tc::fence_after_sync();
-      const uint32_t idesc = tc::idesc_bf16(kTcM, kTcN, 0, 0);
-      for (int ch = 0; ch < nch; ++ch) {
-#pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks)
-          tc::mma_bf16_ss(tbase + SM::cS + ch * kTcN, tc::smem_desc_sw128(qa + (ks / 4) * kTcM * 128 + (ks % 4) * 32, 16, 1024),
-                          tc::smem_desc_sw128(ka + ch * kTcN * D * 2 + (ks / 4) * kTcN * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
-      }
-      tc::mma_commit(&bar[0]);
-    }
-    __syncwarp();
-    if (nxt.pl < dm.SB) load_rows(nxt, pid_s[nbuf]);        // gathers fly while this tile is processed
-    load_pids(nn);
-    store_prev();                                           // the previous tile's rows leave meanwhile
-    float M = -INFINITY, l = 0.f;
-    if (nch > 0) {
-      if (!tc::mbar_wait(&bar[0], ph0)) ok_ = false;
-      ph0 ^= 1;
-      tc::fence_after_sync();
-      // softmax over up to 128 keys: warpgroup = key chunk; the two halves of a row meet through shared memory
-      float sv[kTcN];
-      const int visc = vis - wg * kTcN;                     // visible columns of this warpgroup's chunk
-      float mx = -INFINITY;
-      if (wg < nch) {
-        tc::tmem_ld32(tl + SM::cS + wg * kTcN, *reinterpret_cast<float(*)[32]>(&sv[0]));
-        tc::tmem_ld32(tl + SM::cS + wg * kTcN + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
-#pragma unroll
-        for (int i = 0; i < kTcN; ++i) { sv[i] = i < visc ? sv[i] * scale2 : -INFINITY; mx = fmaxf(mx, sv[i]); }
-      }
-      mx_s[wg][row] = mx;
-      __syncthreads();
-      M = fmaxf(mx_s[0][row], mx_s[1][row]);
-      float rs = 0.f;
-      if (wg < nch) {
-        const float base = M == -INFINITY ? 0.f : M;
-        uint32_t pk[kTcN / 2];
-#pragma unroll
-        for (int i = 0; i < kTcN; i += 2) {
-          __nv_bfloat162 b = __floats2bfloat162_rn(tc::fast_exp2(sv[i] - base), tc::fast_exp2(sv[i + 1] - base));
-          rs += __low2float(b) + __high2float(b);            // the rounded values, as the P V product sees them
-          pk[i / 2] = *reinterpret_cast<uint32_t*>(&b);
+  for (; kc0 < kall || first_sweep; kc0 += kRcKeys, first_sweep = false) {
+    __syncthreads();                                        // the previous sweep is done with the key / value tiles
+    // the cluster's keys (K-major for S = Q K^T) and values (MN-major for O = P V), two chunks of 64
+    if (cw) {
+      for (int ch = 0; ch < 2; ++ch) {
+        const int n = min(kTcN, max(0, kall - kc0 - ch * kTcN));
+        for (int e = tid; e < kTcN * (D / 8); e += kRcCompute) {
+          const int r = e / (D / 8), ck = e % (D / 8);
+          uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
+          if (r < n) {
+            a = reinterpret_cast<const uint4*>(Kb + (size_t)(kc0 + ch * kTcN + r) * D)[ck];
+            b = reinterpret_cast<const uint4*>(Vb + (size_t)(kc0 + ch * kTcN + r) * D)[ck];
+          }
+          const uint32_t off = ch * kTcN * D * 2 + (ck >> 3) * kTcN * 128 + tc::sw128_off(r, ck & 7);
+          *reinterpret_cast<uint4*>(sm + SM::k + off) = a;
+          *reinterpret_cast<uint4*>(sm + SM::v + off) = b;
         }
-#pragma unroll
-        for (int ch8 = 0; ch8 < kTcN / 8; ++ch8)
-          *reinterpret_cast<uint4*>(sm + SM::p + wg * kTcM * kTcN * 2 + tc::sw128_off(row, ch8)) =
-              make_uint4(pk[ch8 * 4], pk[ch8 * 4 + 1], pk[ch8 * 4 + 2], pk[ch8 * 4 + 3]);
       }
-      sum_s[wg][row] = rs;
       tc::fence_async_smem();
-      tc::fence_before_sync();
-      __syncthreads();
-      if (tid == 0) {
-        tc::fence_after_sync();
-        const uint32_t idesc = tc::idesc_bf16(kTcM, D, 0, 1);
-        for (int ch = 0; ch < nch; ++ch) {
+    }
+    Item cur = skip(first_from(0), sub), nxt = next_of(cur), nn = next_of(nxt);
+    load_pids(cur);
+    if (tid < kTcM) { pid_s[0][tid] = pidreg; tok_s[0][tid] = tokreg; }
+    load_pids(nxt);
+    __syncthreads();
+    int buf = 0, qb = 0, tno = 0;                           // slot of the pair-id ring / half of the Q double buffer / tile count
+    if (gw && cur.pl < dm.SB) gather_rows(cur, tok_s[0], 0);
+    bool pre = false;                                       // the logits of the current tile are already issued
+    while (cur.pl < dm.SB) {
+      const int nq = min(kTcM, cur.g1 - cur.t0);
+      const int vis = min(kRcKeys, max(0, ok[cur.pl + 1] - kc0));   // keys of this sweep that the plane sees
+      const int nch = (vis + kTcN - 1) / kTcN;
+      const int nbuf = buf == 2 ? 0 : buf + 1;
+      const int nch_next = chunks_of(nxt);
+      const bool pre_next = nch > 0 && nch_next > 0;        // this tile's last barrier also starts the next tile
+      if (tid < kTcM) { pid_s[nbuf][tid] = pidreg; tok_s[qb ^ 1][tid] = tokreg; }     // ids of the next tile
+      // ids of the next tile visible to the gather warps; the other half of the Q buffer was last read by the
+      // previous tile's logits, which the softmax warps have consumed
+      if (cw || gw) tc::named_bar_sync(1, kRcCompute + kRcGather);
+      if (gw) {
+        if (nxt.pl < dm.SB) gather_rows(nxt, tok_s[qb ^ 1], qb ^ 1);
+        cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf; qb ^= 1;
+        continue;
+      }
+      if (!pre) {
+        // first tile of the sweep, or the tile before had no key chunk: wait for this tile's rows here
+        if (cw) { wait_rows(qb); tc::fence_async_smem(); }
+        sync_cw_issuer();
+        if (tid == kRcIssuer && nch > 0) { tc::fence_after_sync(); issue_s(qb, nch); }
+      }
+      if (cw) load_pids(nn);
+      float M = -INFINITY, l = 0.f;
+      if (nch > 0) {
+        if (cw) {
+          if (ok_ && !tc::mbar_wait(&bar[0], ph0)) ok_ = false;
+          tc::fence_after_sync();
+          // softmax over up to 128 keys: warpgroup = key chunk; the two halves of a row meet through shared memory
+          float sv[kTcN];
+          const int visc = vis - wg * kTcN;                   // visible columns of this warpgroup's chunk
+          float mx = -INFINITY;
+          if (wg < nch) {
+            tc::tmem_ld32(tl + SM::cS + wg * kTcN, *reinterpret_cast<float(*)[32]>(&sv[0]));
+            tc::tmem_ld32(tl + SM::cS + wg * kTcN + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
 #pragma unroll
-          for (int ks = 0; ks < kTcN / 16; ++ks)
-            tc::mma_bf16_ss(tbase + SM::cO, tc::smem_desc_sw128(pa + ch * kTcM * kTcN * 2 + ks * 32, 16, 1024),
-                            tc::smem_desc_sw128(va + ch * kTcN * D * 2 + ks * 16 * 128, kTcN * 128, 1024), idesc, ch > 0 || ks > 0);
+            for (int i = 0; i < kTcN; ++i) { sv[i] = i < visc ? sv[i] * scale2 : -INFINITY; mx = fmaxf(mx, sv[i]); }
+          }
+          mx_s[wg][row] = mx;
+          tc::named_bar_sync(3, kRcCompute);
+          M = fmaxf(mx_s[0][row], mx_s[1][row]);
+          wait_pv();                                          // the previous P V product has read the P tiles
+          float rs = 0.f;
+          if (wg < nch) {
+            const float base = M == -INFINITY ? 0.f : M;
+            uint32_t pk[kTcN / 2];
+#pragma unroll
+            for (int i = 0; i < kTcN; i += 2) {
+              __nv_bfloat162 b = __floats2bfloat162_rn(tc::fast_exp2(sv[i] - base), tc::fast_exp2(sv[i + 1] - base));
+              rs += __low2float(b) + __high2float(b);          // the rounded values, as the P V product sees them
+              pk[i / 2] = *reinterpret_cast<uint32_t*>(&b);
+            }
+#pragma unroll
+            for (int ch8 = 0; ch8 < kTcN / 8; ++ch8)
+              *reinterpret_cast<uint4*>(sm + SM::p + wg * kTcM * kTcN * 2 + tc::sw128_off(row, ch8)) =
+                  make_uint4(pk[ch8 * 4], pk[ch8 * 4 + 1], pk[ch8 * 4 + 2], pk[ch8 * 4 + 3]);
+          }
+          sum_s[wg][row] = rs;
+          if (pre_next) wait_rows(qb ^ 1);                    // the next tile's rows, for the logits issued below
+          tc::fence_async_smem();
         }
-        tc::mma_commit(&bar[1]);
-      }
-      __syncwarp();
-      l = sum_s[0][row] + sum_s[1][row];
-      if (!tc::mbar_wait(&bar[1], ph1)) ok_ = false;
-      ph1 ^= 1;
-      tc::fence_after_sync();
-    }
-    // what the deferred store needs: 1 / l and the log-sum-exp of the row (natural log)
-    prev_inv = l > 0.f ? 1.f / l : 0.f;
-    prev_lse = l > 0.f ? (M + log2f(l)) * 0.6931471805599453f : -INFINITY;
-    prev_nq = nq; prev_buf = buf; pending = true; prev_first = first_sweep;
-    if (nch == 0) {
-      // nothing visible (possible with forced selections): rows of zeros, done here because the accumulator holds no data
-      if (row < nq && ok_) {
-        const size_t pid = (size_t)pq * dm.N * dm.m + pid_s[buf][row];
-        uint4* dst = reinterpret_cast<uint4*>(o_part + pid * D + wg * (D / 2));
+        ph0 ^= 1;
+        sync_cw_issuer();
+        if (tid == kRcIssuer) {
+          tc::fence_after_sync();
+          const uint32_t idesc = tc::idesc_bf16(kTcM, D, 0, 1);
+          for (int ch = 0; ch < nch; ++ch) {
 #pragma unroll
-        for (int i = 0; i < D / 16; ++i) dst[i] = make_uint4(0u, 0u, 0u, 0u);
-        if (wg == 0) l_part[pid] = -INFINITY;
+            for (int ks = 0; ks < kTcN / 16; ++ks)
+              tc::mma_bf16_ss(tbase + SM::cO + (tno & 1) * D, tc::smem_desc_sw128(pa + ch * kTcM * kTcN * 2 + ks * 32, 16, 1024),
+                              tc::smem_desc_sw128(va + ch * kTcN * D * 2 + ks * 16 * 128, kTcN * 128, 1024), idesc, ch > 0 || ks > 0);
+          }
+          tc::mma_commit(&bar[1]);
+          if (pre_next) issue_s(qb ^ 1, nch_next);            // queued behind it: the next tile's logits
+        }
+        if (cw) l = sum_s[0][row] + sum_s[1][row];
       }
-      pending = false;
+      if (cw) {
+        // The previous tile's rows leave now, while the tensor core works (the accumulators alternate).
+        store_prev();
+        pv_pending = nch > 0;                                 // this tile's product, waited for in the next tile
+        // what the deferred store needs: 1 / l and the log-sum-exp of the row (natural log)
+        prev_inv = l > 0.f ? 1.f / l : 0.f;
+        prev_lse = l > 0.f ? (M + log2f(l)) * 0.6931471805599453f : -INFINITY;
+        prev_nq = nq; prev_buf = buf; prev_o = tno & 1; pending = true; prev_first = first_sweep;
+        if (nch == 0) {
+          // nothing visible (possible with forced selections): rows of zeros, done here because the accumulator holds no data
+          if (row < nq && ok_) {
+            const size_t pid = (size_t)pq * dm.N * dm.m + pid_s[buf][row];
+            uint4* dst = reinterpret_cast<uint4*>(o_part + pid * D + wg * (D / 2));
+#pragma unroll
+            for (int i = 0; i < D / 16; ++i) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+            if (wg == 0) l_part[pid] = -INFINITY;
+          }
+          pending = false;
+        }
+      }
+      pre = pre_next;
+      tc::fence_before_sync();
+      cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf; qb ^= 1; ++tno;
     }
-    tc::fence_before_sync();
-    cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf;
-  }
-  store_prev();
+    if (cw) store_prev();
   }
   tc::fence_before_sync();
   __syncthreads();
