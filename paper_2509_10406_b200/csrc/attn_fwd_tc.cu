@@ -471,6 +471,13 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   const float scale2 = dm.sigma * 1.4426950408889634f;
   uint32_t ph0 = 0, ph1 = 0, ph_rows[2] = {0, 0};
   bool ok_ = true;
+#ifdef MUSE_PHASE_CLOCKS
+  long long pc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  const long long t_in_ = clock64();
+#define RCLK(k) { long long n_ = clock64(); pc[k] += n_ - z_; z_ = n_; }
+#else
+#define RCLK(k)
+#endif
   // Every warp walks the same sequence of tiles to the end, whatever happens (after a wait ran out the
   // remaining waits are skipped), so the barriers below always see all their warps.
   auto sync_cw_issuer = [&]() {                            // softmax warps and the issuing warp
@@ -637,6 +644,9 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
     if (gw && cur.pl < dm.SB) gather_rows(cur, tok_s[0], 0);
     bool pre = false;                                       // the logits of the current tile are already issued
     while (cur.pl < dm.SB) {
+#ifdef MUSE_PHASE_CLOCKS
+      long long z_ = clock64();
+#endif
       const int nq = min(kTcM, cur.g1 - cur.t0);
       const int vis = min(kRcKeys, max(0, ok[cur.pl + 1] - kc0));   // keys of this sweep that the plane sees
       const int nch = (vis + kTcN - 1) / kTcN;
@@ -658,47 +668,59 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
         sync_cw_issuer();
         if (tid == kRcIssuer && nch > 0) { tc::fence_after_sync(); issue_s(qb, nch); }
       }
+      RCLK(0)
       if (cw) load_pids(nn);
       float M = -INFINITY, l = 0.f;
       if (nch > 0) {
         if (cw) {
           if (ok_ && !tc::mbar_wait(&bar[0], ph0)) ok_ = false;
           tc::fence_after_sync();
-          // softmax over up to 128 keys: warpgroup = key chunk; the two halves of a row meet through shared memory
-          float sv[kTcN];
-          const int visc = vis - wg * kTcN;                   // visible columns of this warpgroup's chunk
+          RCLK(1)
+          // softmax over up to 128 keys: each warpgroup takes 32 columns of every chunk; the two halves of a row
+          // meet through shared memory.  The logits are read from TMEM twice (row maximum, then probabilities)
+          // rather than kept in registers across the barrier.
           float mx = -INFINITY;
-          if (wg < nch) {
-            tc::tmem_ld32(tl + SM::cS + wg * kTcN, *reinterpret_cast<float(*)[32]>(&sv[0]));
-            tc::tmem_ld32(tl + SM::cS + wg * kTcN + 32, *reinterpret_cast<float(*)[32]>(&sv[32]));
+          for (int ch = 0; ch < nch; ++ch) {
+            float sv[32];
+            tc::tmem_ld32(tl + SM::cS + ch * kTcN + 32 * wg, sv);
+            const int visc = vis - ch * kTcN - 32 * wg;         // visible columns among these 32
 #pragma unroll
-            for (int i = 0; i < kTcN; ++i) { sv[i] = i < visc ? sv[i] * scale2 : -INFINITY; mx = fmaxf(mx, sv[i]); }
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, i < visc ? sv[i] : -INFINITY);
           }
-          mx_s[wg][row] = mx;
+          mx_s[wg][row] = mx * scale2;                          // (scale2 > 0)
+          RCLK(2)
           tc::named_bar_sync(3, kRcCompute);
+          RCLK(3)
           M = fmaxf(mx_s[0][row], mx_s[1][row]);
           wait_pv();                                          // the previous P V product has read the P tiles
           float rs = 0.f;
-          if (wg < nch) {
-            const float base = M == -INFINITY ? 0.f : M;
-            uint32_t pk[kTcN / 2];
+          const float base = M == -INFINITY ? 0.f : M;
+          for (int ch = 0; ch < nch; ++ch) {
+            float sv[32];
+            tc::tmem_ld32(tl + SM::cS + ch * kTcN + 32 * wg, sv);
+            const int visc = vis - ch * kTcN - 32 * wg;
+            uint32_t pk[16];
 #pragma unroll
-            for (int i = 0; i < kTcN; i += 2) {
-              __nv_bfloat162 b = __floats2bfloat162_rn(tc::fast_exp2(sv[i] - base), tc::fast_exp2(sv[i + 1] - base));
+            for (int i = 0; i < 32; i += 2) {
+              const float e0 = i < visc ? tc::fast_exp2(fmaf(sv[i], scale2, -base)) : 0.f;
+              const float e1 = i + 1 < visc ? tc::fast_exp2(fmaf(sv[i + 1], scale2, -base)) : 0.f;
+              __nv_bfloat162 b = __floats2bfloat162_rn(e0, e1);
               rs += __low2float(b) + __high2float(b);          // the rounded values, as the P V product sees them
               pk[i / 2] = *reinterpret_cast<uint32_t*>(&b);
             }
 #pragma unroll
-            for (int ch8 = 0; ch8 < kTcN / 8; ++ch8)
-              *reinterpret_cast<uint4*>(sm + SM::p + wg * kTcM * kTcN * 2 + tc::sw128_off(row, ch8)) =
-                  make_uint4(pk[ch8 * 4], pk[ch8 * 4 + 1], pk[ch8 * 4 + 2], pk[ch8 * 4 + 3]);
+            for (int c4 = 0; c4 < 4; ++c4)
+              *reinterpret_cast<uint4*>(sm + SM::p + ch * kTcM * kTcN * 2 + tc::sw128_off(row, 4 * wg + c4)) =
+                  make_uint4(pk[c4 * 4], pk[c4 * 4 + 1], pk[c4 * 4 + 2], pk[c4 * 4 + 3]);
           }
           sum_s[wg][row] = rs;
+          RCLK(4)
           if (pre_next) wait_rows(qb ^ 1);                    // the next tile's rows, for the logits issued below
           tc::fence_async_smem();
         }
         ph0 ^= 1;
         sync_cw_issuer();
+        RCLK(5)
         if (tid == kRcIssuer) {
           tc::fence_after_sync();
           const uint32_t idesc = tc::idesc_bf16(kTcM, D, 0, 1);
@@ -716,6 +738,10 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
       if (cw) {
         // The previous tile's rows leave now, while the tensor core works (the accumulators alternate).
         store_prev();
+        RCLK(6)
+#ifdef MUSE_PHASE_CLOCKS
+        pc[7] += 1;
+#endif
         pv_pending = nch > 0;                                 // this tile's product, waited for in the next tile
         // what the deferred store needs: 1 / l and the log-sum-exp of the row (natural log)
         prev_inv = l > 0.f ? 1.f / l : 0.f;
@@ -739,6 +765,12 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
     }
     if (cw) store_prev();
   }
+#ifdef MUSE_PHASE_CLOCKS
+  if (tid == 0 && pc[7] >= 12 && atomicCAS(status + 40, 0, 1) == 0) {
+    for (int k = 0; k < 8; ++k) status[41 + k] = (int)pc[k];
+    status[49] = (int)(clock64() - t_in_);
+  }
+#endif
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tbase, SM::cols);
