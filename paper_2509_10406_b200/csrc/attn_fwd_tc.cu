@@ -172,7 +172,7 @@ __device__ __forceinline__ void tc_teardown(TcCtx& c, int tid, int* status) {
 // through shared memory.  Software pipeline over the key tiles t (K and V tiles arrive by TMA):
 //   S(t+1) = Q K_{t+1}^T is issued as soon as S(t) has landed (two S buffers in TMEM, two K tiles in
 //   shared memory), so it runs while the threads do the softmax of tile t; O(t) = P(t) V_t is
-//   collected at the start of iteration t + 1, which frees P and V for tile t + 1.
+//   awaited at the start of iteration t + 1, which frees P and V for tile t + 1; O accumulates in TMEM.
 constexpr int kLfThreads = 256;
 
 template <int D> struct LfSmem {
@@ -247,27 +247,21 @@ k_local_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_k, const __grid_c
   }
   const float scale2 = dm.sigma * 1.4426950408889634f;
   const int my_limit = q0 + row;                            // last visible key of this row
-  float o[HD], m2 = -INFINITY, l = 0.f;                     // l: this warpgroup's share of the row sum
-#pragma unroll
-  for (int i = 0; i < HD; ++i) o[i] = 0.f;
-  auto collect = [&](int t) {                               // O(t) has landed: add this thread's half row
-    if (!tc::mbar_wait(&barPV, t & 1)) ok = false;
-    tc::fence_after_sync();
-#pragma unroll
-    for (int d0 = 0; d0 < HD; d0 += 32) {
-      float v[32];
-      tc::tmem_ld32(tl + cO + wg * HD + d0, v);
-#pragma unroll
-      for (int i = 0; i < 32; ++i) o[d0 + i] += v[i];
-    }
-  };
+  // The output accumulates in TMEM over all key tiles.  m2 is the exponent base in use for this row (log2
+  // units): it follows the running maximum lazily, only when that has grown by more than kLazy (probabilities
+  // then stay below 2^kLazy), and only then is the accumulator rescaled, for every row of the tile at once.
+  constexpr float kLazy = 8.f;
+  float m2 = -INFINITY, l = 0.f;                            // l: this warpgroup's share of the row sum
   for (int t = 0; t < T && ok; ++t) {
     const int c0 = k_lo + t * kTcN, nk = min(kTcN, k_hi - c0);
     if (!tc::mbar_wait(&barS[t & 1], (t >> 1) & 1)) { ok = false; break; }
     tc::fence_after_sync();
     if (tid == 0 && t + 1 < T) issue_s(t + 1);              // runs during this tile's softmax
     __syncwarp();
-    if (t > 0) collect(t - 1);                              // frees P and V (thread 0 has seen the products complete)
+    if (t > 0) {                                            // O(t-1) has landed: P and V are free (thread 0 has seen it too)
+      if (!tc::mbar_wait(&barPV, (t - 1) & 1)) ok = false;
+      tc::fence_after_sync();
+    }
     if (tid == 0) {
       load_v(t);
       if (t + 2 < T) load_k(t + 2);                         // over K_t, which S(t) has consumed
@@ -279,10 +273,26 @@ k_local_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_k, const __grid_c
 #pragma unroll
     for (int i = 0; i < 32; ++i) { s[i] = i < vis ? s[i] * scale2 : -INFINITY; mx = fmaxf(mx, s[i]); }
     mx_s[wg][row] = mx;
-    __syncthreads();
-    const float mn = fmaxf(m2, fmaxf(mx_s[0][row], mx_s[1][row]));
-    const float base = mn == -INFINITY ? 0.f : mn;
-    const float resc = tc::fast_exp2(m2 - base);
+    // (the first tile gives every row a finite maximum: it holds the block's first key)
+    const int grow = __syncthreads_or(t > 0 && mx > m2 + kLazy);
+    const float mt = fmaxf(mx_s[0][row], mx_s[1][row]);
+    if (t == 0) {
+      m2 = mt;
+    } else if (grow) {
+      const float mn = mt > m2 + kLazy ? mt : m2;           // rows that did not grow keep their base (factor 1)
+      const float resc = tc::fast_exp2(m2 - mn);
+#pragma unroll
+      for (int d0 = 0; d0 < HD; d0 += 32) {
+        float v[32];
+        tc::tmem_ld32(tl + cO + wg * HD + d0, v);
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v[i] *= resc;
+        tc::tmem_st32(tl + cO + wg * HD + d0, v);
+      }
+      l *= resc;
+      m2 = mn;
+    }
+    const float base = m2 == -INFINITY ? 0.f : m2;
     float rs = 0.f;
 #pragma unroll
     for (int ch = 0; ch < 4; ++ch) {
@@ -295,12 +305,7 @@ k_local_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_k, const __grid_c
       }
       *reinterpret_cast<uint4*>(Ps + tc::sw128_off(row, 4 * wg + ch)) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
     }
-    l = l * resc + rs;
-    m2 = mn;
-    if (resc != 1.f) {
-#pragma unroll
-      for (int i = 0; i < HD; ++i) o[i] *= resc;
-    }
+    l += rs;
     tc::fence_async_smem();
     tc::fence_before_sync();
     __syncthreads();
@@ -311,24 +316,34 @@ k_local_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_k, const __grid_c
 #pragma unroll
       for (int ks = 0; ks < kTcN / 16; ++ks)
         tc::mma_bf16_ss(tbase + cO, tc::smem_desc_sw128(pa + ks * 32, 16, 1024),
-                        tc::smem_desc_sw128(va + ks * 16 * 128, kTcN * 128, 1024), idesc, ks > 0);
+                        tc::smem_desc_sw128(va + ks * 16 * 128, kTcN * 128, 1024), idesc, t > 0 || ks > 0);
       tc::mma_commit(&barPV);
     }
     __syncwarp();
   }
-  if (ok && T > 0) collect(T - 1);
+  if (ok && T > 0) {
+    if (!tc::mbar_wait(&barPV, (T - 1) & 1)) ok = false;
+    tc::fence_after_sync();
+  }
   // the two halves of the row sum meet
   __syncthreads();
   mx_s[wg][row] = l;
   __syncthreads();
   const float lt = mx_s[0][row] + mx_s[1][row];
-  if (ok && row < nq) {
+  if (ok && T > 0) {
     const size_t t = (size_t)pq * dm.N + q0 + row;
     const float inv = 1.f / lt;
     float4* dst = reinterpret_cast<float4*>(o_loc + t * D + wg * HD);
 #pragma unroll
-    for (int i = 0; i < HD / 4; ++i) dst[i] = make_float4(o[4 * i] * inv, o[4 * i + 1] * inv, o[4 * i + 2] * inv, o[4 * i + 3] * inv);
-    if (wg == 0) lse_loc[t] = (m2 + log2f(lt)) * 0.6931471805599453f;
+    for (int d0 = 0; d0 < HD; d0 += 32) {
+      float v[32];
+      tc::tmem_ld32(tl + cO + wg * HD + d0, v);
+      if (row < nq) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) dst[d0 / 4 + i] = make_float4(v[4 * i] * inv, v[4 * i + 1] * inv, v[4 * i + 2] * inv, v[4 * i + 3] * inv);
+      }
+    }
+    if (wg == 0 && row < nq) lse_loc[t] = (m2 + log2f(lt)) * 0.6931471805599453f;
   }
   tc::fence_before_sync();
   __syncthreads();
