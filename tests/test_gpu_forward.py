@@ -22,6 +22,9 @@ EDGE = {
     # clusters of ~128 keys (several key sweeps in the retrieval kernels)
     "long_segments": CASES["d128"].with_(Hq=1, Hkv=1, N=4096, S=4, Cq=8, Ck=128, m=4),
     "long_clusters": CASES["d128"].with_(Hq=1, Hkv=1, N=4096, S=4, Cq=16, Ck=16, m=4),
+    # four key clusters that every query retrieves: ~48 tiles of 128 pairs per cluster, so that each cluster's
+    # tiles are dealt to several CTAs of the retrieval kernels, and ~2000 keys per cluster (many key sweeps)
+    "shared_clusters": CASES["d128"].with_(Hq=1, Hkv=1, N=8192, S=4, Cq=16, Ck=4, m=4),
 }
 
 
