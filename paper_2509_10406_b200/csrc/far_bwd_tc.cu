@@ -1,4 +1,4 @@
-// Far-field backward on the tensor cores (bf16 mode, D = 128, Ck a multiple of 128, <= 1024).
+// Far-field backward on the tensor cores (bf16 mode, D = 128, Ck a multiple of 128, <= 2048).
 // One CTA per (query cluster i, plane, head) segment.  Clusters sit on the MMA M side (128 per
 // tile, one TMEM lane each), the segment's queries on the N side (64 per sweep; a longer segment
 // takes further sweeps that add to the stored gradients).  Per cluster tile, with L the merged log-sum-exp and delta = dO.O:
@@ -413,7 +413,8 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 }
 
 bool far_bwd_tc_supported(const Dims& d, int dtype) {
-  return dtype == MUSE_BF16 && d.D == fb::D && d.Ck % fb::TJ == 0 && d.Ck <= 1024;
+  // (the far-set mask, 8 bytes per key cluster, shares the CTA's shared memory with 200 KB of tiles)
+  return dtype == MUSE_BF16 && d.D == fb::D && d.Ck % fb::TJ == 0 && d.Ck <= 2048;
 }
 
 int far_bwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const void* dO, const float* qbar, const float* LSE,

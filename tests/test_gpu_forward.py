@@ -25,6 +25,9 @@ EDGE = {
     # four key clusters that every query retrieves: ~48 tiles of 128 pairs per cluster, so that each cluster's
     # tiles are dealt to several CTAs of the retrieval kernels, and ~2000 keys per cluster (many key sweeps)
     "shared_clusters": CASES["d128"].with_(Hq=1, Hkv=1, N=8192, S=4, Cq=16, Ck=4, m=4),
+    # 2048 key clusters: sixteen cluster tiles per segment in the tensor far-field backward (the forward far
+    # field takes its other path above 1024 clusters)
+    "many_key_clusters": CASES["d128"].with_(Hq=1, Hkv=1, N=4096, S=4, Cq=8, Ck=2048, m=4),
 }
 
 
