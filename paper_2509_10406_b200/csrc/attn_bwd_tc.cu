@@ -471,14 +471,21 @@ k_local_bwd_dkdv_tc(Dims dm, const __grid_constant__ CUtensorMap tm_q, const __g
   const int k0 = bstart + kt * kBM, nk = min(kBM, bend - k0);
   const int T = (bend - k0 + kBN - 1) / kBN;                // query tiles that see these keys
   const int u = k0 + row;
-  auto load_scalars = [&](int t) {                          // threads 0..63: L (log2 units) and delta of query tile t
+  // threads 0..63: L (log2 units) and delta of query tile t; loaded into registers one tile before they are
+  // stored, so that no warp waits for global memory in front of a barrier
+  float Lnext = 0.f, dnext = 0.f;
+  auto fetch_scalars = [&](int t) {
     if (tid < kBN && t < T) {
       const int q = k0 + t * kBN + tid;
-      Ls[t % 3][tid] = q < bend ? LSE[(size_t)pq * dm.N + q] * kLog2e : 0.f;
-      ds[t % 3][tid] = q < bend ? delta[(size_t)pq * dm.N + q] : 0.f;
+      Lnext = q < bend ? LSE[(size_t)pq * dm.N + q] * kLog2e : 0.f;
+      dnext = q < bend ? delta[(size_t)pq * dm.N + q] : 0.f;
     }
   };
-  load_scalars(0); load_scalars(1); load_scalars(2);
+  auto store_scalars = [&](int t) {
+    if (tid < kBN && t < T) { Ls[t % 3][tid] = Lnext; ds[t % 3][tid] = dnext; }
+  };
+  fetch_scalars(0); store_scalars(0); fetch_scalars(1); store_scalars(1); fetch_scalars(2); store_scalars(2);
+  fetch_scalars(3);
   tc::fence_before_sync();
   __syncthreads();
   tc::fence_after_sync();
@@ -532,15 +539,17 @@ k_local_bwd_dkdv_tc(Dims dm, const __grid_constant__ CUtensorMap tm_q, const __g
       tc::tmem_ld32(tl + (t & 1) * 2 * kBN + kBN + 32 * wg, dp);
       const float* Lt = Ls[t % 3] + 32 * wg;
       const float* dt = ds[t % 3] + 32 * wg;
+      // bit c of `vis`: query column 32 wg + c exists and sees this thread's key (causal, key inside the tile)
+      const int lo = max(0, u - q0 - 32 * wg), hi = row < nk ? min(32, nq - 32 * wg) : 0;
+      const uint32_t vis = hi > lo ? ((hi >= 32 ? 0xffffffffu : (1u << hi) - 1u) & (lo >= 32 ? 0u : 0xffffffffu << lo)) : 0u;
 #pragma unroll
       for (int k = 0; k < 8; ++k) {
         const float4 a = *reinterpret_cast<const float4*>(Lt + 4 * k), b = *reinterpret_cast<const float4*>(dt + 4 * k);
         const float Lc[4] = {a.x, a.y, a.z, a.w}, dc[4] = {b.x, b.y, b.z, b.w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-          const int col = 32 * wg + 4 * k + e;
-          const float ev = tc::fast_exp2(s[4 * k + e] * scale2 - Lc[e]);
-          const float pv = (col < nq && row < nk && u <= q0 + col) ? ev : 0.f;
+          const float ev = tc::fast_exp2(fmaf(s[4 * k + e], scale2, -Lc[e]));
+          const float pv = (vis >> (4 * k + e)) & 1u ? ev : 0.f;
           p[4 * k + e] = pv;
           g[4 * k + e] = pv * (dp[4 * k + e] - dc[e]);
         }
@@ -550,7 +559,8 @@ k_local_bwd_dkdv_tc(Dims dm, const __grid_constant__ CUtensorMap tm_q, const __g
       if (!tc::mbar_wait(&bar2, (t - 1) & 1)) { ok = false; break; }
       tc::fence_after_sync();
       if (tid == kLdkIssuer && t + 2 < T) load_qd(t + 2);
-      load_scalars(t + 2);
+      store_scalars(t + 2);                                 // fetched during the previous tile
+      fetch_scalars(t + 3);
     }
     if (warp < 8) {
       store_row32(sm + SM::pt, row, wg, p);
