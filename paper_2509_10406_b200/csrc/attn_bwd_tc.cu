@@ -473,16 +473,21 @@ k_local_bwd_dkdv_tc(Dims dm, const __grid_constant__ CUtensorMap tm_q, const __g
   const int u = k0 + row;
   // threads 0..63: L (log2 units) and delta of query tile t; loaded into registers one tile before they are
   // stored, so that no warp waits for global memory in front of a barrier
+  // (nothing may depend on the loaded values before store_scalars: a dependent instruction placed earlier
+  // would make these warps wait for global memory)
   float Lnext = 0.f, dnext = 0.f;
   auto fetch_scalars = [&](int t) {
     if (tid < kBN && t < T) {
-      const int q = k0 + t * kBN + tid;
-      Lnext = q < bend ? LSE[(size_t)pq * dm.N + q] * kLog2e : 0.f;
-      dnext = q < bend ? delta[(size_t)pq * dm.N + q] : 0.f;
+      const int q = min(k0 + t * kBN + tid, bend - 1);
+      Lnext = LSE[(size_t)pq * dm.N + q];
+      dnext = delta[(size_t)pq * dm.N + q];
     }
   };
   auto store_scalars = [&](int t) {
-    if (tid < kBN && t < T) { Ls[t % 3][tid] = Lnext; ds[t % 3][tid] = dnext; }
+    if (tid < kBN && t < T) {
+      const bool in = k0 + t * kBN + tid < bend;
+      Ls[t % 3][tid] = in ? Lnext * kLog2e : 0.f; ds[t % 3][tid] = in ? dnext : 0.f;
+    }
   };
   fetch_scalars(0); store_scalars(0); fetch_scalars(1); store_scalars(1); fetch_scalars(2); store_scalars(2);
   fetch_scalars(3);
@@ -526,63 +531,76 @@ k_local_bwd_dkdv_tc(Dims dm, const __grid_constant__ CUtensorMap tm_q, const __g
     issue1(0);
   }
   const float scale2 = dm.sigma * kLog2e;
-  for (int t = 0; t < T && ok; ++t) {
-    const int q0 = k0 + t * kBN, nq = min(kBN, bend - q0);
-    if (!tc::mbar_wait(&bar1[t & 1], (t >> 1) & 1)) { ok = false; break; }
-    tc::fence_after_sync();
-    if (tid == kLdkIssuer && t + 1 < T) issue1(t + 1);       // runs while this tile's P^T, G^T are computed
-    __syncwarp();
-    float p[32], g[32];
-    if (warp < 8) {
-      float s[32], dp[32];
-      tc::tmem_ld32(tl + (t & 1) * 2 * kBN + 32 * wg, s);
-      tc::tmem_ld32(tl + (t & 1) * 2 * kBN + kBN + 32 * wg, dp);
-      const float* Lt = Ls[t % 3] + 32 * wg;
-      const float* dt = ds[t % 3] + 32 * wg;
-      // bit c of `vis`: query column 32 wg + c exists and sees this thread's key (causal, key inside the tile)
-      const int lo = max(0, u - q0 - 32 * wg), hi = row < nk ? min(32, nq - 32 * wg) : 0;
-      const uint32_t vis = hi > lo ? ((hi >= 32 ? 0xffffffffu : (1u << hi) - 1u) & (lo >= 32 ? 0u : 0xffffffffu << lo)) : 0u;
-#pragma unroll
-      for (int k = 0; k < 8; ++k) {
-        const float4 a = *reinterpret_cast<const float4*>(Lt + 4 * k), b = *reinterpret_cast<const float4*>(dt + 4 * k);
-        const float Lc[4] = {a.x, a.y, a.z, a.w}, dc[4] = {b.x, b.y, b.z, b.w};
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const float ev = tc::fast_exp2(fmaf(s[4 * k + e], scale2, -Lc[e]));
-          const float pv = (vis >> (4 * k + e)) & 1u ? ev : 0.f;
-          p[4 * k + e] = pv;
-          g[4 * k + e] = pv * (dp[4 * k + e] - dc[e]);
+  // Two loops over the query tiles, one per role, that meet at one CTA-wide barrier per tile (P^T / G^T
+  // written).  Each role's instructions are contiguous: no warp jumps over the other role's code.  Every warp
+  // runs all T tiles whatever happens (after a wait ran out the remaining waits are skipped).
+  if (warp == 8) {
+    for (int t = 0; t < T; ++t) {
+      if (tid == kLdkIssuer) {
+        if (t + 1 < T) issue1(t + 1);                       // its accumulator buffer was read before the last barrier
+        if (t > 0) {                                        // MMA2(t - 1) has completed: its ring slot is free
+          if (ok && !tc::mbar_wait(&bar2, (t - 1) & 1)) ok = false;
+          if (t + 2 < T) load_qd(t + 2);
         }
       }
+      tc::fence_before_sync();
+      __syncthreads();
+      if (tid == kLdkIssuer) {
+        tc::fence_after_sync();
+        const uint32_t qa = tc::smem_u32(sm + SM::qd + (t % 3) * SM::tile), da = qa + kBN * D * 2;
+        const uint32_t idesc = tc::idesc_bf16(kBM, D, 0, 1);
+#pragma unroll
+        for (int ks = 0; ks < kBN / 16; ++ks)
+          tc::mma_bf16_ss(tbase + SM::cDV, tc::smem_desc_sw128(pa + ks * 32, 16, 1024), desc_mn<kBN>(da, ks), idesc, t > 0 || ks > 0);
+#pragma unroll
+        for (int ks = 0; ks < kBN / 16; ++ks)
+          tc::mma_bf16_ss(tbase + SM::cDK, tc::smem_desc_sw128(ga + ks * 32, 16, 1024), desc_mn<kBN>(qa, ks), idesc, t > 0 || ks > 0);
+        tc::mma_commit(&bar2);
+      }
+      __syncwarp();
     }
-    if (t > 0) {                                            // MMA2(t - 1) has completed: P^T / G^T and its ring slot are free
-      if (!tc::mbar_wait(&bar2, (t - 1) & 1)) { ok = false; break; }
+  } else {
+    for (int t = 0; t < T; ++t) {
+      const int q0 = k0 + t * kBN, nq = min(kBN, bend - q0);
+      if (ok && !tc::mbar_wait(&bar1[t & 1], (t >> 1) & 1)) ok = false;
       tc::fence_after_sync();
-      if (tid == kLdkIssuer && t + 2 < T) load_qd(t + 2);
-      store_scalars(t + 2);                                 // fetched during the previous tile
-      fetch_scalars(t + 3);
-    }
-    if (warp < 8) {
+      float p[32], g[32];
+      {
+        float s[32], dp[32];
+        tc::tmem_ld32(tl + (t & 1) * 2 * kBN + 32 * wg, s);
+        tc::tmem_ld32(tl + (t & 1) * 2 * kBN + kBN + 32 * wg, dp);
+        const float* Lt = Ls[t % 3] + 32 * wg;
+        const float* dt = ds[t % 3] + 32 * wg;
+        // bit c of `vis`: query column 32 wg + c exists and sees this thread's key (causal, key inside the tile)
+        const int lo = max(0, u - q0 - 32 * wg), hi = row < nk ? min(32, nq - 32 * wg) : 0;
+        const uint32_t vis = hi > lo ? ((hi >= 32 ? 0xffffffffu : (1u << hi) - 1u) & (lo >= 32 ? 0u : 0xffffffffu << lo)) : 0u;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+          const float4 a = *reinterpret_cast<const float4*>(Lt + 4 * k), b = *reinterpret_cast<const float4*>(dt + 4 * k);
+          const float Lc[4] = {a.x, a.y, a.z, a.w}, dc[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const float ev = tc::fast_exp2(fmaf(s[4 * k + e], scale2, -Lc[e]));
+            const float pv = (vis >> (4 * k + e)) & 1u ? ev : 0.f;
+            p[4 * k + e] = pv;
+            g[4 * k + e] = pv * (dp[4 * k + e] - dc[e]);
+          }
+        }
+      }
+      if (t > 0) {                                          // MMA2(t - 1) has completed: P^T / G^T are free
+        if (ok && !tc::mbar_wait(&bar2, (t - 1) & 1)) ok = false;
+        tc::fence_after_sync();
+        store_scalars(t + 2);                               // fetched during the previous tile
+        fetch_scalars(t + 3);
+      }
       store_row32(sm + SM::pt, row, wg, p);
       store_row32(sm + SM::gt, row, wg, g);
+      tc::fence_async_smem();
+      tc::fence_before_sync();
+      __syncthreads();
     }
-    tc::fence_async_smem();
-    tc::fence_before_sync();
-    __syncthreads();
-    if (tid == kLdkIssuer) {
-      tc::fence_after_sync();
-      const uint32_t qa = tc::smem_u32(sm + SM::qd + (t % 3) * SM::tile), da = qa + kBN * D * 2;
-      const uint32_t idesc = tc::idesc_bf16(kBM, D, 0, 1);
-#pragma unroll
-      for (int ks = 0; ks < kBN / 16; ++ks)
-        tc::mma_bf16_ss(tbase + SM::cDV, tc::smem_desc_sw128(pa + ks * 32, 16, 1024), desc_mn<kBN>(da, ks), idesc, t > 0 || ks > 0);
-#pragma unroll
-      for (int ks = 0; ks < kBN / 16; ++ks)
-        tc::mma_bf16_ss(tbase + SM::cDK, tc::smem_desc_sw128(ga + ks * 32, 16, 1024), desc_mn<kBN>(qa, ks), idesc, t > 0 || ks > 0);
-      tc::mma_commit(&bar2);
-    }
-    __syncwarp();
   }
+  ok = __syncthreads_and(ok);
   if (ok && T > 0) { if (!tc::mbar_wait(&bar2, (T - 1) & 1)) ok = false; }
   tc::fence_after_sync();
   if (warp < 8) {                                           // warpgroup 0 writes dV, warpgroup 1 writes dK (all their threads run the TMEM loads)
