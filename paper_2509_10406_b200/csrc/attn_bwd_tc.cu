@@ -507,15 +507,23 @@ k_local_bwd_dkdv_tc(Dims dm, const __grid_constant__ CUtensorMap tm_q, const __g
       tc::tma_load_2d(slot + kBN * D * 2 + g * kBN * 128, &tm_do, 64 * g, r, &barQ[t % 3]);
     }
   };
+  // one descriptor per operand buffer, stepped per MMA (K-major views; the MN-major views of the ring differ in lbo)
+  const uint64_t dk0 = tc::smem_desc_sw128(ka, 16, 1024), dv0 = tc::smem_desc_sw128(va, 16, 1024),
+                 dq0 = tc::smem_desc_sw128(tc::smem_u32(sm + SM::qd), 16, 1024),
+                 dqm0 = tc::smem_desc_sw128(tc::smem_u32(sm + SM::qd), kBN * 128, 1024),
+                 dp0 = tc::smem_desc_sw128(pa, 16, 1024), dg0 = tc::smem_desc_sw128(ga, 16, 1024);
   auto issue1 = [&](int t) {                                // S^T(t) = K Q_t^T, dP^T(t) = V dO_t^T into accumulator buffer t & 1
     if (!tc::mbar_wait(&barQ[t % 3], (t / 3) & 1)) ok = false;
     tc::fence_after_sync();
-    const uint32_t qa = tc::smem_u32(sm + SM::qd + (t % 3) * SM::tile), da = qa + kBN * D * 2;
+    const uint32_t slot = (uint32_t)(t % 3) * SM::tile;
     const uint32_t idesc = tc::idesc_bf16(kBM, kBN, 0, 0), cb = tbase + (t & 1) * 2 * kBN;
+    const uint64_t qd = tc::desc_step(dq0, slot), dd = tc::desc_step(dq0, slot + kBN * D * 2);
 #pragma unroll
-    for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(cb, desc_k<kBM>(ka, ks), desc_k<kBN>(qa, ks), idesc, ks > 0);
+    for (int ks = 0; ks < D / 16; ++ks)
+      tc::mma_bf16_ss(cb, tc::desc_step(dk0, (ks / 4) * kBM * 128 + (ks % 4) * 32), tc::desc_step(qd, (ks / 4) * kBN * 128 + (ks % 4) * 32), idesc, ks > 0);
 #pragma unroll
-    for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(cb + kBN, desc_k<kBM>(va, ks), desc_k<kBN>(da, ks), idesc, ks > 0);
+    for (int ks = 0; ks < D / 16; ++ks)
+      tc::mma_bf16_ss(cb + kBN, tc::desc_step(dv0, (ks / 4) * kBM * 128 + (ks % 4) * 32), tc::desc_step(dd, (ks / 4) * kBN * 128 + (ks % 4) * 32), idesc, ks > 0);
     tc::mma_commit(&bar1[t & 1]);
   };
   if (tid == kLdkIssuer) {
@@ -547,14 +555,16 @@ k_local_bwd_dkdv_tc(Dims dm, const __grid_constant__ CUtensorMap tm_q, const __g
       __syncthreads();
       if (tid == kLdkIssuer) {
         tc::fence_after_sync();
-        const uint32_t qa = tc::smem_u32(sm + SM::qd + (t % 3) * SM::tile), da = qa + kBN * D * 2;
+        const uint32_t slot = (uint32_t)(t % 3) * SM::tile;
         const uint32_t idesc = tc::idesc_bf16(kBM, D, 0, 1);
+        const uint64_t qm = tc::desc_step(dqm0, slot), dm_ = tc::desc_step(dqm0, slot + kBN * D * 2);
+        const uint32_t acc = t > 0;
 #pragma unroll
         for (int ks = 0; ks < kBN / 16; ++ks)
-          tc::mma_bf16_ss(tbase + SM::cDV, tc::smem_desc_sw128(pa + ks * 32, 16, 1024), desc_mn<kBN>(da, ks), idesc, t > 0 || ks > 0);
+          tc::mma_bf16_ss(tbase + SM::cDV, tc::desc_step(dp0, ks * 32), tc::desc_step(dm_, ks * 16 * 128), idesc, ks > 0 ? 1u : acc);
 #pragma unroll
         for (int ks = 0; ks < kBN / 16; ++ks)
-          tc::mma_bf16_ss(tbase + SM::cDK, tc::smem_desc_sw128(ga + ks * 32, 16, 1024), desc_mn<kBN>(qa, ks), idesc, t > 0 || ks > 0);
+          tc::mma_bf16_ss(tbase + SM::cDK, tc::desc_step(dg0, ks * 32), tc::desc_step(qm, ks * 16 * 128), idesc, ks > 0 ? 1u : acc);
         tc::mma_commit(&bar2);
       }
       __syncwarp();

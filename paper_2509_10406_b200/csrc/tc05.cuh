@@ -108,6 +108,10 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
   d |= 2ull << 61;          // SWIZZLE_128B
   return d;
 }
+// The descriptor of the same layout `byte_off` bytes further on (the start address sits in the low 14 bits in
+// 16-byte units; shared-memory addresses stay below 256 KB, so the sum never carries out of the field).
+// Kernels build one descriptor per operand buffer and step it with this: one add per MMA in the issuing thread.
+__device__ __forceinline__ uint64_t desc_step(uint64_t d, uint32_t byte_off) { return d + (uint64_t)(byte_off >> 4); }
 // Instruction descriptor for kind::f16 with bf16 inputs and fp32 accumulation.
 __host__ __device__ constexpr uint32_t idesc_bf16(int M, int N, int a_mn_major, int b_mn_major) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
