@@ -1,4 +1,4 @@
-// Far-field forward on the tensor cores (bf16 mode, D = 128, Ck a multiple of 128, Ck <= 1024).
+// Far-field forward on the tensor cores (bf16 mode, D = 128, Ck a multiple of 128, Ck <= 2048).
 // One CTA per (query cluster i, plane, head) segment; its queries (32 on average at the headline
 // sizes, up to 64 per pass) share the Ck accumulated summaries of (i, plane).  The summaries sit
 // on the MMA M side (128 clusters per tile, one TMEM lane each) and the queries on the N side
@@ -21,7 +21,9 @@ typedef __nv_bfloat16 bf16;
 int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
 
 constexpr int kFD = 128, kFJ = 128;                 // head dim, clusters per tile
-constexpr int kFR = 64, kFQ = 16;                   // queries per pass, queries per selection step
+// Queries per pass FR and per selection step FQ (one warp each) are template parameters: 64 / 16 up to 1024
+// key clusters, 32 / 8 up to 2048 (all FR x Ck scores of a pass live in the 512 TMEM columns, P and the score
+// rows of a step in shared memory).
 constexpr int kTileBytes = kFJ * kFD * 2;           // 32 KB: one [128][128] bf16 operand tile
 constexpr int kFarTcCols = 512;
 constexpr int kMaxStA = 6, kMaxStD = 4;
@@ -29,21 +31,21 @@ constexpr int kCandMax = 128;                       // candidates kept by the co
 
 struct FarBars { uint64_t fullA[kMaxStA], emptyA[kMaxStA], fullD[kMaxStD], emptyD[kMaxStD], done; };
 
-constexpr int kFarTcThreads = 512;      // 16 warps: one query each in the selection steps
 
-// Top-m of one query's scores s[0..Ck) (one warp; Ck <= 1024).  Writes the chosen clusters to
+// Top-m of one query's scores s[0..Ck) (one warp; Ck <= 32 NKMAX).  Writes the chosen clusters to
 // so[0..m) (-1 padded), and removes them from the far set by setting their score to -inf.
 // Order-preserving integer keys; the key T of the m-th largest is found by bisection with warp
 // reductions, everything above T is taken and, among ties at T, the lowest cluster indices.
 // When few scores can reach the top m (bounded below by the m-th largest lane maximum), they are
 // first compacted into `cand` (kCandMax keys then kCandMax indices, 128-byte segments `seg`
 // bytes apart) so that every bisection round touches 4 keys per lane instead of Ck / 32.
+template <int NKMAX>
 __device__ __forceinline__ void select_top_m(float* s, int Ck, int m, int32_t* so, int lane, unsigned char* cand, int seg,
                                              bool may_compact) {
-  const int NK = Ck >> 5;                       // scores per lane (<= 32)
-  uint32_t key[32];
+  const int NK = Ck >> 5;                       // scores per lane (<= NKMAX)
+  uint32_t key[NKMAX];
 #pragma unroll
-  for (int k = 0; k < 32; ++k) {
+  for (int k = 0; k < NKMAX; ++k) {
     const uint32_t b = __float_as_uint(k < NK ? s[lane + 32 * k] : -INFINITY);
     key[k] = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
   }
@@ -52,14 +54,14 @@ __device__ __forceinline__ void select_top_m(float* s, int Ck, int m, int32_t* s
   auto count_ge = [&](uint32_t thr) {           // lane-local count, then one warp reduction
     int c = 0;
 #pragma unroll
-    for (int k = 0; k < 32; ++k) c += key[k] >= thr ? 1 : 0;
+    for (int k = 0; k < NKMAX; ++k) c += key[k] >= thr ? 1 : 0;
     return (int)__reduce_add_sync(0xffffffffu, (unsigned)c);
   };
   // lane-local statistics in one sweep: finite count, largest and second largest key, smallest finite key
   uint32_t m1 = 0u, m2 = 0u, kmn = 0xffffffffu;
   int nfin = 0;
 #pragma unroll
-  for (int k = 0; k < 32; ++k) {
+  for (int k = 0; k < NKMAX; ++k) {
     m2 = max(m2, min(m1, key[k]));
     m1 = max(m1, key[k]);
     const bool fin = key[k] >= kFinite;
@@ -95,7 +97,7 @@ __device__ __forceinline__ void select_top_m(float* s, int Ck, int m, int32_t* s
     if (compacted) {
       int base = 0;
 #pragma unroll
-      for (int k = 0; k < 32; ++k) {
+      for (int k = 0; k < NKMAX; ++k) {
         if (k < NK) {
           const bool in = key[k] >= kmn;
           const uint32_t mb = __ballot_sync(0xffffffffu, in);
@@ -145,7 +147,7 @@ __device__ __forceinline__ void select_top_m(float* s, int Ck, int m, int32_t* s
   } else {
     const int need = take_all ? 0 : m - count_ge(T + 1u);
 #pragma unroll
-    for (int k = 0; k < 32; ++k) {
+    for (int k = 0; k < NKMAX; ++k) {
       if (k < NK) {
         const bool tie = !take_all && key[k] == T;
         const bool gt = take_all ? key[k] >= kFinite : key[k] > T;
@@ -161,17 +163,19 @@ __device__ __forceinline__ void select_top_m(float* s, int Ck, int m, int32_t* s
   for (int k = base + lane; k < m; k += 32) so[k] = -1;
 }
 
-__global__ void __launch_bounds__(kFarTcThreads, 1)
+template <int FR, int FQ>
+__global__ void __launch_bounds__(FQ * 32, 1)
 k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_constant__ CUtensorMap tm_klo,
              const __grid_constant__ CUtensorMap tm_nu, const bf16* __restrict__ Q, const int32_t* __restrict__ off_q,
              const int32_t* __restrict__ perm_q, const float* __restrict__ mu, const float* __restrict__ beta,
              const int32_t* __restrict__ sel_in, int32_t* __restrict__ sel_out, float* __restrict__ o_far,
              float* __restrict__ lse_far, int p_bytes, int sc_bytes, int nsA, int nsD, int* __restrict__ status) {
+  constexpr int NT = FQ * 32, NTG = FQ / 4, KT = 16 / NTG;   // threads; tile groups in the TMEM read-out; cluster tiles per group
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ FarBars bars;
   __shared__ uint32_t tbase_s;
-  __shared__ int32_t rows[kFR];
-  __shared__ float rinv[kFR];
+  __shared__ int32_t rows[FR];
+  __shared__ float rinv[FR];
   __shared__ int32_t selq[kMaxM];
   const int i = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z;
   const int blk = dm.causal ? pl + 1 : 0, Ck = dm.Ck, NJ = Ck / kFJ, m = dm.m;
@@ -224,18 +228,18 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   bool ok = true;
   const int lq = warp & 3, tg = warp >> 2;            // TMEM lane quarter of this warp, tile group
 
-  for (int r0 = p0; r0 < p1 && ok; r0 += kFR) {
-    const int n = min(kFR, p1 - r0);
+  for (int r0 = p0; r0 < p1 && ok; r0 += FR) {
+    const int n = min(FR, p1 - r0);
 #ifdef MUSE_PHASE_CLOCKS
     long long ck0 = clock64(), ck1 = 0, ck3 = 0, ck4 = 0;
 #endif
-    if (tid < kFR) rows[tid] = tid < n ? pm[r0 + tid] : -1;
+    if (tid < FR) rows[tid] = tid < n ? pm[r0 + tid] : -1;
     // query rows -> K-major swizzled tile [64][128] bf16 (2 blocks of [64][128 B])
-    for (int e = tid; e < kFR * (kFD / 8); e += kFarTcThreads) {
+    for (int e = tid; e < FR * (kFD / 8); e += NT) {
       const int r = e >> 4, ck = e & 15, kb = ck >> 3, c = ck & 7;
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
       if (r < n) v = reinterpret_cast<const uint4*>(Qp + (size_t)pm[r0 + r] * kFD)[ck];
-      *reinterpret_cast<uint4*>(Qs + kb * kFR * 128 + tc::sw128_off(r, c)) = v;
+      *reinterpret_cast<uint4*>(Qs + kb * FR * 128 + tc::sw128_off(r, c)) = v;
     }
     tc::fence_async_smem();
     tc::fence_before_sync();
@@ -260,7 +264,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       }
     } else if (tid == 32) {
       tc::fence_after_sync();
-      const uint32_t idesc = tc::idesc_bf16(kFJ, kFR, 0, 0);
+      const uint32_t idesc = tc::idesc_bf16(kFJ, FR, 0, 0);
       const uint32_t qa = tc::smem_u32(Qs);
       const int T = 2 * NJ;
       for (int u = 0; u < T; ++u, ++cntA) {
@@ -270,15 +274,15 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
         const uint32_t a0 = tc::smem_u32(sm + s * kTileBytes);
 #pragma unroll
         for (int ks = 0; ks < kFD / 16; ++ks)
-          tc::mma_bf16_ss(tbase + (u >> 1) * kFR, tc::smem_desc_sw128(a0 + (ks / 4) * kFJ * 128 + (ks % 4) * 32, 16, 1024),
-                          tc::smem_desc_sw128(qa + (ks / 4) * kFR * 128 + (ks % 4) * 32, 16, 1024), idesc, (u & 1) || ks > 0);
+          tc::mma_bf16_ss(tbase + (u >> 1) * FR, tc::smem_desc_sw128(a0 + (ks / 4) * kFJ * 128 + (ks % 4) * 32, 16, 1024),
+                          tc::smem_desc_sw128(qa + (ks / 4) * FR * 128 + (ks % 4) * 32, 16, 1024), idesc, (u & 1) || ks > 0);
         tc::mma_commit(&bars.emptyA[s]);
       }
       if (ok) tc::mma_commit(&bars.done);
     }
-    float bq[2];                                        // beta of this thread's clusters, loaded ahead of the TMEM reads
+    float bq[KT];                                       // beta of this thread's clusters, loaded ahead of the TMEM reads
 #pragma unroll
-    for (int k = 0; k < 2; ++k) { const int jt = tg + 4 * k; bq[k] = jt < NJ ? bep[jt * kFJ + (tid & 127)] : 0.f; }
+    for (int k = 0; k < KT; ++k) { const int jt = tg + NTG * k; bq[k] = jt < NJ ? bep[jt * kFJ + (tid & 127)] : 0.f; }
     __syncwarp();     // lanes 1..31 of warp 0 park here instead of spinning beside the issuing lane
     if (!tc::mbar_wait(&bars.done, done_ph)) ok = false;
     done_ph ^= 1;
@@ -286,28 +290,29 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #ifdef MUSE_PHASE_CLOCKS
     ck1 = clock64();
 #endif
-    for (int qs = 0; qs * kFQ < n; ++qs) {
+    for (int qs = 0; qs * FQ < n; ++qs) {
       // ---- B: TMEM -> sc[r][j] for the 16 queries of this step
 #ifdef MUSE_PHASE_CLOCKS
       long long cb0 = clock64(), cb1 = 0, cb2 = 0, cb3 = 0;
 #endif
 #pragma unroll
-      for (int k = 0; k < 2; ++k) {
-        const int jt = tg + 4 * k;
+      for (int k = 0; k < KT; ++k) {
+        const int jt = tg + NTG * k;
         if (jt >= NJ) break;
-        float v[16];
-        tc::tmem_ld16(tbase + ((uint32_t)(lq * 32) << 16) + jt * kFR + qs * kFQ, v);
+        float v[FQ];
+        if constexpr (FQ == 16) tc::tmem_ld16(tbase + ((uint32_t)(lq * 32) << 16) + jt * FR + qs * FQ, v);
+        else tc::tmem_ld8(tbase + ((uint32_t)(lq * 32) << 16) + jt * FR + qs * FQ, v);
         const int j = jt * kFJ + (tid & 127);
         const float b = bq[k];
 #pragma unroll
-        for (int r = 0; r < kFQ; ++r) sc[r * Ck + j] = b == -INFINITY ? -INFINITY : fmaf(v[r], dm.sigma, b);
+        for (int r = 0; r < FQ; ++r) sc[r * Ck + j] = b == -INFINITY ? -INFINITY : fmaf(v[r], dm.sigma, b);
       }
       __syncthreads();
 #ifdef MUSE_PHASE_CLOCKS
       cb1 = clock64();
 #endif
       // ---- C: selection + softmax of the far set; P (bf16) as a K-major operand [64][Ck]
-      const int r = qs * kFQ + warp;                    // one query per warp
+      const int r = qs * FQ + warp;                    // one query per warp
       float* s = sc + warp * Ck;
       float sum = 0.f, mx = -INFINITY;
       if (r < n) {
@@ -320,7 +325,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
           for (int k = lane; k < m; k += 32) { int c = selq[k]; so[k] = c; if (c >= 0) s[c] = -INFINITY; }
         } else if (m > 0) {
           // this query's own (not yet written) P row doubles as the candidate scratch
-          select_top_m(s, Ck, m, so, lane, Pm + r * 128, kFR * 128, Ck >= 512);
+          select_top_m<(FR == 64 ? 32 : 64)>(s, Ck, m, so, lane, Pm + r * 128, FR * 128, Ck >= 512);
         }
         __syncwarp();
 #ifdef MUSE_PHASE_CLOCKS
@@ -342,7 +347,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
           sum += __low2float(b) + __high2float(b);
           w[k] = *reinterpret_cast<uint32_t*>(&b);
         }
-        *reinterpret_cast<uint4*>(Pm + (q >> 3) * (kFR * 128) + tc::sw128_off(r, q & 7)) = make_uint4(w[0], w[1], w[2], w[3]);
+        *reinterpret_cast<uint4*>(Pm + (q >> 3) * (FR * 128) + tc::sw128_off(r, q & 7)) = make_uint4(w[0], w[1], w[2], w[3]);
       }
       sum = warp_sum(sum);
       if (lane == 0) {
@@ -376,7 +381,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       }
     } else if (tid == 32 && ok) {
       tc::fence_after_sync();
-      const uint32_t idesc = tc::idesc_bf16(kFD, kFR, 1, 0);
+      const uint32_t idesc = tc::idesc_bf16(kFD, FR, 1, 0);
       const uint32_t pa = tc::smem_u32(Pm);
       unsigned char* ring = sm + p_bytes;
       for (int u = 0; u < NJ; ++u, ++cntD) {
@@ -387,7 +392,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #pragma unroll
         for (int ks = 0; ks < kFJ / 16; ++ks)
           tc::mma_bf16_ss(tbase, tc::smem_desc_sw128(a0 + ks * 16 * 128, kFJ * 128, 1024),
-                          tc::smem_desc_sw128(pa + (2 * u + ks / 4) * (kFR * 128) + (ks % 4) * 32, 16, 1024), idesc,
+                          tc::smem_desc_sw128(pa + (2 * u + ks / 4) * (FR * 128) + (ks % 4) * 32, 16, 1024), idesc,
                           u > 0 || ks > 0);
         tc::mma_commit(&bars.emptyD[s]);
       }
@@ -405,7 +410,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     }
 #endif
     // ---- E: thread = output dim d; warps 0-3 read queries 0..31, warps 4-7 queries 32..63
-    if (warp < 8) {
+    if (warp < FR / 8) {
       const int half = warp >> 2;
       float v[32];
       tc::tmem_ld32(tbase + ((uint32_t)(lq * 32) << 16) + 32 * half, v);
@@ -425,7 +430,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 }
 
 bool far_fwd_tc_supported(const Dims& d, int dtype) {
-  return dtype == MUSE_BF16 && d.D == kFD && d.Ck % kFJ == 0 && d.Ck <= 1024 && d.Ck >= kFJ;
+  return dtype == MUSE_BF16 && d.D == kFD && d.Ck % kFJ == 0 && d.Ck <= 2048 && d.Ck >= kFJ;
 }
 
 int far_fwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const int32_t* off_q, const int32_t* perm_q,
@@ -436,17 +441,25 @@ int far_fwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const int32_t* 
   if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&klo, sp.klo, ent, kFD, kFJ);
   if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&nu, sp.nu, ent, kFD, kFJ);
   if (rc != MUSE_OK) return rc;
-  const int p_bytes = kFR * d.Ck * 2;                                   // P: bf16 [64][Ck]
-  int sc_bytes = kFQ * d.Ck * 4;                                        // 16 score rows, later the nu ring
+  const bool wide = d.Ck > 1024;                                         // 32 queries per pass, 8 per selection step
+  const int FR = wide ? 32 : 64, FQ = wide ? 8 : 16;
+  const int p_bytes = FR * d.Ck * 2;                                     // P: bf16 [FR][Ck]
+  int sc_bytes = FQ * d.Ck * 4;                                          // FQ score rows, later the nu ring
   if (sc_bytes < 2 * kTileBytes) sc_bytes = 2 * kTileBytes;
   int nsA = (p_bytes + sc_bytes) / kTileBytes, nsD = sc_bytes / kTileBytes;
   nsA = nsA > kMaxStA ? kMaxStA : nsA;
   nsD = nsD > kMaxStD ? kMaxStD : nsD;
-  const size_t smem = (size_t)p_bytes + sc_bytes + kFR * kFD * 2 + 1024;
-  MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_fwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const size_t smem = (size_t)p_bytes + sc_bytes + FR * kFD * 2 + 1024;
   prof_mark("k_far_fwd_tc", st);
-  k_far_fwd_tc<<<dim3(d.Cq, d.SB, d.B * d.Hq), kFarTcThreads, smem, st>>>(d, khi, klo, nu, (const bf16*)Q, off_q, perm_q, sp.mu, sp.beta,
-                                                               sel_in, sel_out, o_far, lse_far, p_bytes, sc_bytes, nsA, nsD, status);
+  if (wide) {
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_fwd_tc<32, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k_far_fwd_tc<32, 8><<<dim3(d.Cq, d.SB, d.B * d.Hq), 256, smem, st>>>(d, khi, klo, nu, (const bf16*)Q, off_q, perm_q, sp.mu, sp.beta,
+                                                                 sel_in, sel_out, o_far, lse_far, p_bytes, sc_bytes, nsA, nsD, status);
+  } else {
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_fwd_tc<64, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k_far_fwd_tc<64, 16><<<dim3(d.Cq, d.SB, d.B * d.Hq), 512, smem, st>>>(d, khi, klo, nu, (const bf16*)Q, off_q, perm_q, sp.mu, sp.beta,
+                                                                   sel_in, sel_out, o_far, lse_far, p_bytes, sc_bytes, nsA, nsD, status);
+  }
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }
