@@ -235,6 +235,7 @@ def main():
     ap.add_argument("--impl", default="muse", choices=["muse", "reference"])
     ap.add_argument("--gain", type=float, default=1.0, help="multiplier on Q (1 = literal workload)")
     ap.add_argument("--m", type=int, default=None, help="override retrieved clusters per query")
+    ap.add_argument("--kmeans-iters", type=int, default=None, help="override the number of Lloyd iterations T")
     ap.add_argument("--heads", type=int, default=None, help="override head count (smaller captures)")
     ap.add_argument("--head-groups", type=int, default=0,
                     help="run the KV-head groups in this many sequential stages over one set of buffers "
@@ -255,6 +256,8 @@ def main():
     if args.dipole:
         w = w.with_(m=0)
         args.forward_only = True
+    if args.kmeans_iters is not None:
+        w = w.with_(T=args.kmeans_iters)
     if args.heads is not None:
         w = w.with_(Hq=args.heads, Hkv=max(1, args.heads * w.Hkv // w.Hq))
     if args.impl == "reference":
@@ -299,17 +302,27 @@ def main():
     O_all = torch.empty_like(Q)
     dQ_all, dK_all, dV_all = (None, None, None) if args.forward_only else (torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V))
 
-    def step():
+    marks = []                                            # (stage, event) pairs of the timed steps, when asked for
+
+    def step(mark=False):
+        def m_(name):
+            if mark:
+                e = torch.cuda.Event(enable_timing=True); e.record(); marks.append((name, e))
+        m_("start")
         for g in range(groups):
             qs, ks = slice(g * hq, (g + 1) * hq), slice(g * hkv, (g + 1) * hkv)
             Qg, Kg, Vg = Q[:, qs], K[:, ks], V[:, ks]
             mb.muse_cluster(p, Qg, Kg, init_q[:, qs], init_k[:, ks], buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, buf.ws)
+            m_("cluster")
             mb.muse_summarize(p, Kg, Vg, buf.assign_k, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
+            m_("summarize")
             mb.muse_attn_fwd(p, Qg, Kg, Vg, buf.assign_q, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, None,
                              O_all[:, qs], buf.LSE, buf.sel, buf.ws)
+            m_("forward")
             if not args.forward_only:
                 mb.muse_attn_bwd(p, Qg, Kg, Vg, O_all[:, qs], buf.LSE, dO[:, qs], buf.assign_q, buf.qbar, buf.off_k,
                                  buf.perm_k, buf.summaries, buf.sel, dQ_all[:, qs], dK_all[:, ks], dV_all[:, ks], buf.ws)
+                m_("backward")
 
     def barrier():
         if world > 1:
@@ -328,10 +341,20 @@ def main():
     barrier()
     ev0.record()
     for _ in range(args.steps):
-        step()
+        step(mark=True)
     ev1.record()
     barrier()
     ms = ev0.elapsed_time(ev1) / args.steps
+    # per public call and per step, from events recorded between the calls of the timed steps
+    stages, per_step, t_step = {}, [], 0.0
+    for (n0, e0), (n1, e1) in zip(marks, marks[1:]):
+        if n1 == "start":
+            per_step.append(t_step); t_step = 0.0
+            continue
+        dt = e0.elapsed_time(e1)
+        stages[n1] = stages.get(n1, 0.0) + dt / args.steps
+        t_step += dt
+    per_step.append(t_step)
     prof = mb.muse_profile_report()
     mb.muse_profile(False)
     clocks = sampler.stop() if rank == 0 else None
@@ -504,6 +527,7 @@ def main():
             "data": "synthetic",
             "config": dict(workload_config(w, args.gain), head_stages=groups,
                            dipole=int(args.dipole), passes="cluster+summarize+forward" if args.forward_only else "cluster+summarize+forward+backward"),
+            "ms_per_step_median": statistics.median(per_step), "ms_per_step_best": min(per_step), "stages_ms": stages,
             "clocks": clocks, "e2e": e2e,
             "gpu_launches": launches, "roofline": roof, "cpu_baseline": cpu, "kernels": kernels, "context": context}
     print(json.dumps(line))
