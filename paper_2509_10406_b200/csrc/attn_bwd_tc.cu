@@ -968,7 +968,7 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
 #pragma unroll
               for (int e = 0; e < 4; ++e) a2[e] = __floats2bfloat162_rn(__low2float(a2[e]) + __low2float(o2[e]), __high2float(a2[e]) + __high2float(o2[e]));
             }
-            __stcs(dst, val);
+            *dst = val;
           }
         }
       }

@@ -623,7 +623,7 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
             for (int e = 0; e < 4; ++e)
               a2[e] = __floats2bfloat162_rn(wn * __low2float(a2[e]) + wo * __low2float(o2[e]), wn * __high2float(a2[e]) + wo * __high2float(o2[e]));
           }
-          __stcs(dst, val);
+          *dst = val;
         }
       }
     }
