@@ -32,7 +32,7 @@ UNIT = "tokens/s"
 
 
 # ------------------------------------------------------------------------------------------
-# work models: algorithmic FLOPs / bytes per step for each kernel ("Kernels")
+# work models: algorithmic FLOPs / bytes per step for each kernel
 # ------------------------------------------------------------------------------------------
 def work_model(w: wl.Workload):
     B, Hq, Hkv, N, D, Cq, Ck, m, S, T = w.B, w.Hq, w.Hkv, w.N, w.D, w.Cq, w.Ck, w.m, w.S, w.T
