@@ -19,8 +19,10 @@ Readings taken where the paper is silent (listed again in the design notes):
  * clustering: T Lloyd iterations (assign, update) from given start points,
    then a final assignment against the last centres; qbar := those centres.
    Empty clusters keep their centre; ties go to the lowest index.
- * spatial selection k_2 = all causally visible blocks, so the merge has three
-   non-empty components (far approximation, retrieved exact, local exact).
+ * spatial selection k_2 = all causally visible blocks on the hot path, so the merge has three
+   non-empty components (far approximation, retrieved exact, local exact).  forward(k2 > 0)
+   also states the two-level retrieval (block selection with per-block summaries and the
+   fourth, near-field component); block ties go to the lower block index.  Forward only.
  * top-m: among clusters with at least one visible key, largest score first,
    ties to the lower cluster index; fewer than m candidates -> take them all.
 
@@ -30,7 +32,9 @@ summaries; m = C_k, singleton key clusters or singleton query clusters give
 dense causal softmax attention (textbook formula written separately in the
 test); key-translation invariance; weights sum to one and are causal;
 error bilinear in the residuals; backward vs central finite differences and,
-for m = C_k, vs the closed-form dense-attention gradient.  Dipole: the Jacobian
+for m = C_k, vs the closed-form dense-attention gradient.  Two-level retrieval: k2 >= S - 1
+reproduces k2 = all; a separately written single softmax over exact and stand-in keys on tiny
+inputs; singleton key or query clusters stay exact for every k2; weights causal, sum to one.  Dipole: the Jacobian
 of the far field at zero residual equals the dense-attention Jacobian (a
 cross-covariance written separately in the test), the error falls from first
 to second order in the residual, causality and key-translation invariance.
@@ -291,10 +295,24 @@ def _softmax_part(logits, values):
     return p @ values, lse
 
 
+def select_blocks(bl, k2):
+    """Top-k2 spatial blocks of one (query, selected cluster) pair.  `bl` [nb] are the logits of
+    the per-block summaries (-inf: no visible key of the cluster in that block).  Largest first,
+    ties to the lower block index, fewer than k2 candidates -> all of them.  int32 [k2], -1 padded."""
+    out = np.full(k2, -1, np.int32)
+    order = np.argsort(-bl, kind="stable")
+    cand = order[np.isfinite(bl[order])][:k2]
+    out[:cand.size] = cand
+    return out
+
+
 def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs, m, causal,
-             sel_rows, sel_mode, cbar_ib=None):
+             sel_rows, sel_mode, cbar_ib=None, k2=0, blk_i=None, bsel_rows=None):
     """All quantities of Algorithm 1's per-query loop for the queries `rows`, which share the
-    query cluster (centroid qbar_i) and the spatial block b."""
+    query cluster (centroid qbar_i) and the spatial block b.
+    k2 > 0 (Section "Two-Level Retrieval", spatial block selection): inside every selected cluster
+    only the k2 best-scoring earlier blocks are retrieved exactly; its other earlier blocks enter
+    through their PER-BLOCK summaries `blk_i` = (mu, kappa, nu)[b', j] of this query cluster."""
     N = K.shape[0]
     Ck = muh_ib.shape[0]
     qp = sigma * Q[rows]                                   # full (scaled) query
@@ -326,6 +344,35 @@ def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs
     u = np.arange(N)
     vis = (u // Bs < b) if causal else np.ones(N, bool)
     ret_mask = vis[None, :] & selmask[:, a_k]
+    o_near = np.zeros((len(rows), V.shape[1])); lse_near = np.full(len(rows), -np.inf)
+    bsel = None
+    if k2 > 0 and causal:
+        # 2. block selection inside the selected clusters, with the pre-accumulation summaries
+        mu_b, ka_b, nu_b = blk_i                           # [S, Ck], [S, Ck, D], [S, Ck, Dv]
+        bsel = np.full((len(rows), max(m, 1), k2), -1, np.int32)
+        blk_of = u // Bs
+        ret_mask = np.zeros((len(rows), N), bool)
+        for r in range(len(rows)):
+            near_logits, near_values = [], []
+            for k, j in enumerate(sel_rows[r]):
+                if j < 0:
+                    continue
+                bl = np.full(b, -np.inf)
+                for bp in range(b):                        # block-index causal mask: b' < b
+                    if np.isfinite(mu_b[bp, j]):
+                        bl[bp] = qres[r] @ ka_b[bp, j] + mu_b[bp, j]
+                chosen = select_blocks(bl, k2) if bsel_rows is None else np.asarray(bsel_rows[r][k], np.int32)
+                bsel[r, k] = chosen
+                for bp in range(b):
+                    if not np.isfinite(bl[bp]):
+                        continue
+                    if bp in chosen[chosen >= 0]:
+                        ret_mask[r] |= (a_k == j) & (blk_of == bp)
+                    else:                                  # not retrieved: its per-block summary stands in
+                        near_logits.append(bl[bp]); near_values.append(nu_b[bp, j])
+            if near_logits:
+                o1, l1 = _softmax_part(np.asarray(near_logits)[None, :], np.asarray(near_values))
+                o_near[r], lse_near[r] = o1[0], l1[0]
     logit = qp @ K.T
     ret_logit = np.where(ret_mask, logit, -np.inf)
     o_ret, lse_ret = _softmax_part(ret_logit, V)
@@ -336,12 +383,12 @@ def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs
         loc_mask = np.zeros((len(rows), N), bool)
     loc_logit = np.where(loc_mask, logit, -np.inf)
     o_loc, lse_loc = _softmax_part(loc_logit, V)
-    # merge by log-sum-exp weights (component 2 is empty because k_2 = all)
-    lses = np.stack([lse_far, lse_ret, lse_loc], 1)
+    # merge by log-sum-exp weights (component 2, the near field, is empty when k_2 = all)
+    lses = np.stack([lse_far, lse_ret, lse_loc, lse_near], 1)
     L = _lse(lses, 1)
     wts = np.exp(lses - L[:, None])
-    O = wts[:, 0:1] * o_far + wts[:, 1:2] * o_ret + wts[:, 2:3] * o_loc
-    return dict(O=O, L=L, sel=sel_rows, sel_gap=gap, selmask=selmask, score=score, qp=qp, qres=qres,
+    O = wts[:, 0:1] * o_far + wts[:, 1:2] * o_ret + wts[:, 2:3] * o_loc + wts[:, 3:4] * o_near
+    return dict(O=O, L=L, sel=sel_rows, bsel=bsel, o_near=o_near, lse_near=lse_near, sel_gap=gap, selmask=selmask, score=score, qp=qp, qres=qres,
                 far_logit=far_logit, exact_logit=np.where(ret_mask | loc_mask, logit, -np.inf),
                 o_far=o_far, lse_far=lse_far, o_ret=o_ret, lse_ret=lse_ret,
                 o_loc=o_loc, lse_loc=lse_loc)
@@ -358,14 +405,20 @@ def _segments(a_q, N, S, causal, rows):
 
 
 def forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, sel_mode=0,
-            summ=None, rows=None, dipole=0):
+            summ=None, rows=None, dipole=0, k2=0, bsel=None, blocks=None):
     """MuSe attention for one head.  Returns a dict with O [N,Dv], LSE [N], sel [N,m] and the
     three component (o, lse) pairs.  `sel` forces the retrieved clusters (teacher forcing);
     `rows` restricts the computation to some queries (others are left zero / -inf / -1).
     `dipole=1` adds the untilted pre-merged dipole correction to the far field; the paper
-    defines it without retrieval, so it requires m = 0."""
+    defines it without retrieval, so it requires m = 0.
+    `k2` > 0: two-level retrieval; per (query, selected cluster) only the k2 best earlier blocks
+    are retrieved exactly (returned as bsel [N, m, k2], -1 padded; `bsel` forces them), the other
+    earlier blocks of the selected clusters are approximated by their per-block summaries
+    (`blocks` = block_summaries(...) may be passed in).  k2 = 0 retrieves every visible block."""
     if dipole and m != 0:
         raise ValueError("the dipole correction is defined for m = 0 (no retrieval)")
+    if k2 < 0 or (k2 > 0 and dipole):
+        raise ValueError("k2 must be >= 0 and is not combined with the dipole correction")
     Q = np.asarray(Q, np.float64); K = np.asarray(K, np.float64); V = np.asarray(V, np.float64)
     qbar = np.asarray(qbar, np.float64)
     N, D = Q.shape; Dv = V.shape[1]
@@ -375,22 +428,30 @@ def forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, 
     if summ is None:
         summ = accumulated_summaries(K, V, a_k, qbar, sigma, S, Ck, causal)
     muh, kah, nuh = summ
+    if k2 > 0 and causal and blocks is None:
+        blocks = block_summaries(K, V, a_k, qbar, sigma, S, Ck)
     cbar = merged_dipole(muh, untilted_covariances(K, V, a_k, S, Ck, causal)) if dipole else None
     out = dict(O=np.zeros((N, Dv)), LSE=np.full(N, -np.inf), sel=np.full((N, m), -1, np.int32),
                sel_gap=np.full(N, np.inf))
-    for name in ("o_far", "o_ret", "o_loc"):
+    for name in ("o_far", "o_ret", "o_loc", "o_near"):
         out[name] = np.zeros((N, Dv))
-    for name in ("lse_far", "lse_ret", "lse_loc"):
+    for name in ("lse_far", "lse_ret", "lse_loc", "lse_near"):
         out[name] = np.full(N, -np.inf)
+    if k2 > 0:
+        out["bsel"] = np.full((N, max(m, 1), k2), -1, np.int32)
     for b, i, r in _segments(a_q, N, S, causal, rows):
         seg = _segment(Q, K, V, a_k, qbar[i], muh[b, i], kah[b, i], nuh[b, i], r, b,
                        sigma=sigma, Bs=Bs, m=m, causal=causal,
                        sel_rows=None if sel is None else sel[r], sel_mode=sel_mode,
-                       cbar_ib=None if cbar is None else cbar[b, i])
+                       cbar_ib=None if cbar is None else cbar[b, i], k2=k2,
+                       blk_i=None if blocks is None else (blocks[0][:, i], blocks[1][:, i], blocks[2][:, i]),
+                       bsel_rows=None if bsel is None else bsel[r])
         out["O"][r], out["LSE"][r], out["sel"][r] = seg["O"], seg["L"], seg["sel"]
         out["sel_gap"][r] = seg["sel_gap"]
-        for name in ("o_far", "lse_far", "o_ret", "lse_ret", "o_loc", "lse_loc"):
+        for name in ("o_far", "lse_far", "o_ret", "lse_ret", "o_loc", "lse_loc", "o_near", "lse_near"):
             out[name][r] = seg[name]
+        if k2 > 0 and seg["bsel"] is not None:
+            out["bsel"][r] = seg["bsel"]
     out["summ"] = summ
     out["cbar"] = cbar
     return out
