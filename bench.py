@@ -42,7 +42,7 @@ def work_model(w: wl.Workload):
     nd = N * D
     ret_keys = m * (N / Ck) * (S - 1) / (2 * S)             # nominal retrieved keys per query
     local = 2 * D * N * Bs                                  # 2 matmuls over the causal half
-    far_tc = w.dtype == "bf16" and D == 128 and Ck % 128 == 0 and Ck <= 1024      # tensor-core far-field path
+    far_tc = w.dtype == "bf16" and D == 128 and Ck % 128 == 0 and Ck <= 2048      # tensor-core far-field path
     summ = heads * SB * Cq * Ck * ((3 * D * 2 + 8) if far_tc else (2 * D + 1) * 4)  # accumulated summaries
     grads = heads * SB * Cq * Ck * ((2 * D * 2 + 4) if far_tc else (2 * D + 1) * 4) # their gradients
     part = heads * N * m * D * (2 if w.dtype == "bf16" else 4)                       # retrieval partials (o or dq)
