@@ -836,14 +836,15 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   const uint32_t tl = c.tbase + ((uint32_t)((warp & 3) * 32) << 16);
   const float scale2 = dm.sigma * kLog2e;
 
-  // work items: (plane, first pair of the tile); a plane takes part in a sweep if it has pairs and, from the
-  // second sweep on, if it sees keys of that sweep
+  // work items: (plane, first pair of the tile).  A tile belongs to the same CTA in every sweep (its position
+  // among ALL tiles of the cluster decides), because later sweeps add to the dQ rows that the first one stored;
+  // from the second sweep on, the tiles of planes that see no key of the sweep are passed over.
   struct Item { int pl, t0, g1; };
   for (int kc0 = k0; kc0 < kall || kc0 == k0; kc0 += KC) {
     const bool first_sweep = kc0 == k0;
     auto plane_active = [&](int pl) {
       const int g0 = go[(size_t)pl * dm.Ck], g1 = go[(size_t)pl * dm.Ck + 1];
-      return g1 > g0 && (first_sweep || ok[pl + 1] > kc0);
+      return g1 > g0;
     };
     auto first_from = [&](int pl) {
       Item it; it.pl = pl;
@@ -857,7 +858,9 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       return first_from(a.pl + 1);
     };
     auto skip = [&](Item a, int n) { for (int k = 0; k < n; ++k) a = next1(a); return a; };
-    auto next_of = [&](const Item& a) { return skip(a, nsub); };         // this CTA's next tile
+    auto live = [&](const Item& a) { return a.pl >= dm.SB || first_sweep || ok[a.pl + 1] > kc0; };
+    auto next_of = [&](Item a) { do { a = skip(a, nsub); } while (!live(a)); return a; };   // this CTA's next tile
+    auto first_of = [&]() { Item a = skip(first_from(0), sub); while (!live(a)) a = skip(a, nsub); return a; };
     auto chunks_of = [&](const Item& a) {                                 // key chunks of this sweep that the tile's plane sees
       return a.pl < dm.SB ? (min(KC, max(0, ok[a.pl + 1] - kc0)) + kBN - 1) / kBN : 0;
     };
@@ -916,7 +919,7 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase + SM::cDP, desc_k<kBM>(dab, ks), desc_k<kBN>(vac, ks), idesc, ks > 0);
       tc::mma_commit(&c.bar[0]);
     };
-    Item cur = skip(first_from(0), sub), nxt = next_of(cur), nn = next_of(nxt);
+    Item cur = first_of(), nxt = next_of(cur), nn = next_of(nxt);
     load_pids(cur);
     if (tid < kBM) { pid_s[0][tid] = pidreg; tok_s[0][tid] = tokreg; }
     load_pids(nxt);

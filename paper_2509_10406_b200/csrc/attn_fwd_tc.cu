@@ -511,7 +511,7 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   bool first_sweep = true;
   auto first_from = [&](int pl) {
     Item it; it.pl = pl; it.t0 = 0; it.g1 = 0;
-    while (it.pl < dm.SB && (go[(size_t)it.pl * dm.Ck + 1] <= go[(size_t)it.pl * dm.Ck] || (!first_sweep && ok[it.pl + 1] <= kc0))) ++it.pl;
+    while (it.pl < dm.SB && go[(size_t)it.pl * dm.Ck + 1] <= go[(size_t)it.pl * dm.Ck]) ++it.pl;
     if (it.pl < dm.SB) { it.t0 = go[(size_t)it.pl * dm.Ck]; it.g1 = go[(size_t)it.pl * dm.Ck + 1]; }
     return it;
   };
@@ -521,7 +521,12 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
     return first_from(a.pl + 1);
   };
   auto skip = [&](Item a, int n) { for (int k = 0; k < n; ++k) a = next1(a); return a; };
-  auto next_of = [&](const Item& a) { return skip(a, nsub); };           // this CTA's next tile
+  // A tile belongs to the same CTA in every sweep (its position among ALL tiles of the cluster decides),
+  // because later sweeps add to the rows that the first one stored; from the second sweep on, the
+  // tiles of planes that see no key of the sweep are passed over.
+  auto live = [&](const Item& a) { return a.pl >= dm.SB || first_sweep || ok[a.pl + 1] > kc0; };
+  auto next_of = [&](Item a) { do { a = skip(a, nsub); } while (!live(a)); return a; };   // this CTA's next tile
+  auto first_of = [&]() { Item a = skip(first_from(0), sub); while (!live(a)) a = skip(a, nsub); return a; };
   auto chunks_of = [&](const Item& a) {                                   // key chunks of this sweep that the tile's plane sees
     return a.pl < dm.SB ? (min(kRcKeys, max(0, ok[a.pl + 1] - kc0)) + kTcN - 1) / kTcN : 0;
   };
@@ -650,7 +655,7 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
       }
       tc::fence_async_smem();
     }
-    Item cur = skip(first_from(0), sub), nxt = next_of(cur), nn = next_of(nxt);
+    Item cur = first_of(), nxt = next_of(cur), nn = next_of(nxt);
     load_pids(cur);
     if (tid < kTcM) { pid_s[0][tid] = pidreg; tok_s[0][tid] = tokreg; }
     load_pids(nxt);
