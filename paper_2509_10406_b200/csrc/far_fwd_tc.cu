@@ -33,131 +33,190 @@ struct FarBars { uint64_t fullA[kMaxStA], emptyA[kMaxStA], fullD[kMaxStD], empty
 
 
 // Top-m of one query's scores s[0..Ck) (one warp; Ck <= 32 NKMAX).  Writes the chosen clusters to
-// so[0..m) (-1 padded), and removes them from the far set by setting their score to -inf.
-// Order-preserving integer keys; the key T of the m-th largest is found by bisection with warp
-// reductions, everything above T is taken and, among ties at T, the lowest cluster indices.
-// When few scores can reach the top m (bounded below by the m-th largest lane maximum), they are
-// first compacted into `cand` (kCandMax keys then kCandMax indices, 128-byte segments `seg`
-// bytes apart) so that every bisection round touches 4 keys per lane instead of Ck / 32.
+// so[0..m) (-1 padded, in no particular order), and removes them from the far set by setting
+// their score to -inf.  Scores become order-preserving integer keys; everything above the key T
+// of the m-th largest is taken and, among ties at T, the lowest cluster indices.
+//
+// Fast path (m <= 64, `may_compact`): the m-th largest of the 64 per-lane top-two keys, found by a
+// bitonic sort across the warp (two keys per lane, shuffles only), bounds the m-th largest score
+// from below, and on random data only about m + 4 scores reach it.  Those candidates are
+// compacted into `cand` (kCandMax keys then kCandMax indices, 128-byte segments `seg` bytes apart;
+// a lane-prefix sum gives every lane its slots, so the scatter needs no votes) and T is found by
+// bisection over 4 keys per lane.  The code is laid out for instruction-level parallelism: a
+// warp's chain of dependent votes and reductions, not the issue rate, bounds the selection.
+// General path (any m, many equal scores, fewer than m finite scores): bisection over all keys.
 template <int NKMAX>
 __device__ __forceinline__ void select_top_m(float* s, int Ck, int m, int32_t* so, int lane, unsigned char* cand, int seg,
-                                             bool may_compact) {
+                                             bool may_compact, int* dbg = nullptr) {
+#ifdef MUSE_PHASE_CLOCKS
+  long long c0_ = clock64(), c1_ = 0, c2_ = 0, c3_ = 0, c4_ = 0;
+#define MUSE_SEL_CLOCK(x) x = clock64()
+#else
+#define MUSE_SEL_CLOCK(x)
+#endif
   const int NK = Ck >> 5;                       // scores per lane (<= NKMAX)
-  uint32_t key[NKMAX];
+  auto to_key = [](float x) {
+    const uint32_t b = __float_as_uint(x);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+  };
+  float v[NKMAX];
 #pragma unroll
-  for (int k = 0; k < NKMAX; ++k) {
-    const uint32_t b = __float_as_uint(k < NK ? s[lane + 32 * k] : -INFINITY);
-    key[k] = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-  }
+  for (int k = 0; k < NKMAX; ++k) v[k] = k < NK ? s[lane + 32 * k] : -INFINITY;
   const uint32_t kFinite = 0x00800000u;         // smallest key above key(-inf) = 0x007fffff
   const uint32_t lt = (1u << lane) - 1u;
+  float f1 = -INFINITY, f2 = -INFINITY;         // the lane's largest and second largest score
+#pragma unroll
+  for (int k = 0; k < NKMAX; ++k) {
+    f2 = fmaxf(f2, fminf(f1, v[k]));
+    f1 = fmaxf(f1, v[k]);
+  }
+  const uint32_t m1 = to_key(f1), m2 = to_key(f2);
+  MUSE_SEL_CLOCK(c1_);
+  if (may_compact && m >= 1 && m <= 64) {
+    // bitonic sort, descending, of the 64 keys e = 2 lane + r held as (v0, v1)
+    uint32_t v0 = m1, v1 = m2;
+    const int e2 = lane << 1;
+#pragma unroll
+    for (int k = 2; k <= 64; k <<= 1) {
+      const bool desc = (e2 & k) == 0;
+#pragma unroll
+      for (int j = k >> 1; j >= 2; j >>= 1) {
+        const uint32_t p0 = __shfl_xor_sync(0xffffffffu, v0, j >> 1), p1 = __shfl_xor_sync(0xffffffffu, v1, j >> 1);
+        const bool keep_max = ((e2 & j) == 0) == desc;
+        v0 = keep_max ? max(v0, p0) : min(v0, p0);
+        v1 = keep_max ? max(v1, p1) : min(v1, p1);
+      }
+      const uint32_t hi = max(v0, v1), lo = min(v0, v1);
+      v0 = desc ? hi : lo;
+      v1 = desc ? lo : hi;
+    }
+    const uint32_t lb = __shfl_sync(0xffffffffu, ((m - 1) & 1) ? v1 : v0, (m - 1) >> 1);
+    const uint32_t kmx = __shfl_sync(0xffffffffu, v0, 0);
+    MUSE_SEL_CLOCK(c2_);
+    uint32_t msk[(NKMAX + 31) / 32] = {};                     // this lane's candidates, one bit per score
+    // (float comparison: the same set as by key, plus -0 beside +0, which does no harm)
+    const uint32_t lbb = (lb & 0x80000000u) ? (lb & 0x7fffffffu) : ~lb;
+    const float lbf = __uint_as_float(lbb);
+#pragma unroll
+    for (int k = 0; k < NKMAX; ++k) msk[k >> 5] |= v[k] >= lbf ? 1u << (k & 31) : 0u;
+    int cl = 0;
+#pragma unroll
+    for (int w = 0; w < (NKMAX + 31) / 32; ++w) cl += __popc(msk[w]);
+    int incl = cl;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, incl, d);
+      if (lane >= d) incl += t;
+    }
+    const int ncand = __shfl_sync(0xffffffffu, incl, 31);
+    if (lb >= kFinite && ncand <= kCandMax) {
+      // a lane holds one or two candidates as a rule: walk its mask and fetch the scores again
+      int pos = incl - cl;
+#pragma unroll
+      for (int w = 0; w < (NKMAX + 31) / 32; ++w) {
+        for (uint32_t mm = msk[w]; mm != 0u; mm &= mm - 1u, ++pos) {
+          const int j = lane + 32 * (32 * w + __ffs((int)mm) - 1);
+          *reinterpret_cast<uint32_t*>(cand + (pos >> 5) * seg + (pos & 31) * 4) = to_key(s[j]);
+          *reinterpret_cast<int32_t*>(cand + (4 + (pos >> 5)) * seg + (pos & 31) * 4) = j;
+        }
+      }
+      __syncwarp();
+      MUSE_SEL_CLOCK(c3_);
+      uint32_t ck[4];
+      int32_t ci[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const bool in = lane + 32 * q < ncand;
+        ck[q] = in ? *reinterpret_cast<const uint32_t*>(cand + q * seg + lane * 4) : 0u;
+        ci[q] = in ? *reinterpret_cast<const int32_t*>(cand + (4 + q) * seg + lane * 4) : 0x7fffffff;
+      }
+      auto count4 = [&](uint32_t thr) {
+        return (int)__reduce_add_sync(0xffffffffu, (unsigned)((ck[0] >= thr) + (ck[1] >= thr) + (ck[2] >= thr) + (ck[3] >= thr)));
+      };
+      const int shared = __clz((int)(kmx ^ lb));              // 32 if the interval is a single key
+      uint32_t T = shared >= 32 ? kmx : (kmx & ~(0xffffffffu >> shared));
+      for (int bit = 31 - shared; bit >= 0; --bit) {
+        const uint32_t c2 = T | (1u << bit);
+        const int c = count4(c2);
+        if (c >= m) { T = c2; if (c == m) break; }
+      }
+      MUSE_SEL_CLOCK(c4_);
+#ifdef MUSE_PHASE_CLOCKS
+      if (dbg && lane == 0) { dbg[0] = (int)(c1_ - c0_); dbg[1] = (int)(c2_ - c1_); dbg[2] = (int)(c3_ - c2_); dbg[3] = (int)(c4_ - c3_); dbg[4] = ncand; dbg[5] = 1; }
+#endif
+      int need = m - count4(T + 1u);                            // ties at T still to take (>= 0)
+      const int ntie = (int)__reduce_add_sync(0xffffffffu, (unsigned)((ck[0] == T) + (ck[1] == T) + (ck[2] == T) + (ck[3] == T)));
+      bool take[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) take[q] = ck[q] > T || (ntie <= need && ck[q] == T);
+      if (ntie > need) {
+        // more ties than places: lowest cluster indices first
+        for (; need > 0; --need) {
+          int jm = 0x7fffffff;
+#pragma unroll
+          for (int q = 0; q < 4; ++q) jm = min(jm, (ck[q] == T && !take[q]) ? ci[q] : 0x7fffffff);
+          jm = __reduce_min_sync(0xffffffffu, jm);
+#pragma unroll
+          for (int q = 0; q < 4; ++q) take[q] = take[q] || (ck[q] == T && ci[q] == jm);
+        }
+      }
+      int base = 0;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (32 * q < ncand) {
+          const uint32_t ms = __ballot_sync(0xffffffffu, take[q]);
+          if (take[q]) { so[base + __popc(ms & lt)] = ci[q]; s[ci[q]] = -INFINITY; }
+          base += __popc(ms);
+        }
+      }
+      for (int k = base + lane; k < m; k += 32) so[k] = -1;
+      return;
+    }
+  }
+
+  uint32_t key[NKMAX];
+#pragma unroll
+  for (int k = 0; k < NKMAX; ++k) key[k] = to_key(v[k]);
   auto count_ge = [&](uint32_t thr) {           // lane-local count, then one warp reduction
     int c = 0;
 #pragma unroll
     for (int k = 0; k < NKMAX; ++k) c += key[k] >= thr ? 1 : 0;
     return (int)__reduce_add_sync(0xffffffffu, (unsigned)c);
   };
-  // lane-local statistics in one sweep: finite count, largest and second largest key, smallest finite key
-  uint32_t m1 = 0u, m2 = 0u, kmn = 0xffffffffu;
+  uint32_t kmn = 0xffffffffu;                   // smallest finite key
   int nfin = 0;
 #pragma unroll
   for (int k = 0; k < NKMAX; ++k) {
-    m2 = max(m2, min(m1, key[k]));
-    m1 = max(m1, key[k]);
     const bool fin = key[k] >= kFinite;
     nfin += fin ? 1 : 0;
     kmn = min(kmn, fin ? key[k] : 0xffffffffu);
   }
   const bool take_all = (int)__reduce_add_sync(0xffffffffu, (unsigned)nfin) <= m;
   uint32_t T = kFinite;
-  bool compacted = false;
-  int ncand = 0;
-  uint32_t ck[4] = {0u, 0u, 0u, 0u};
   if (!take_all) {
     const uint32_t kmx = __reduce_max_sync(0xffffffffu, m1);
     kmn = __reduce_min_sync(0xffffffffu, kmn);
-    if (m <= 64) {
-      // the m-th largest of the 64 per-lane top-two keys bounds the m-th largest score from below
-      // (tightly: about m + 4 scores reach it on random data), by bisection over the bits below
-      // the prefix shared by the largest and the smallest finite key
-      const int sh0 = __clz((int)(kmx ^ kmn));
-      uint32_t lb = sh0 >= 32 ? kmx : (kmx & ~(0xffffffffu >> sh0));
-      for (int bit = 31 - sh0; bit >= 0; --bit) {
-        const uint32_t c2 = lb | (1u << bit);
-        if ((int)__reduce_add_sync(0xffffffffu, (unsigned)((m1 >= c2) + (m2 >= c2))) >= m) lb = c2;
-      }
-      kmn = max(kmn, lb);
-      if (may_compact) {
-        ncand = count_ge(kmn);
-        compacted = ncand <= kCandMax;
-      }
-    }
     const int shared = __clz((int)(kmx ^ kmn));            // 32 if the interval is a single key
     T = shared >= 32 ? kmx : (kmx & ~(0xffffffffu >> shared));
-    if (compacted) {
-      int base = 0;
-#pragma unroll
-      for (int k = 0; k < NKMAX; ++k) {
-        if (k < NK) {
-          const bool in = key[k] >= kmn;
-          const uint32_t mb = __ballot_sync(0xffffffffu, in);
-          if (in) {
-            const int pos = base + __popc(mb & lt);
-            *reinterpret_cast<uint32_t*>(cand + (pos >> 5) * seg + (pos & 31) * 4) = key[k];
-            *reinterpret_cast<int32_t*>(cand + (4 + (pos >> 5)) * seg + (pos & 31) * 4) = lane + 32 * k;
-          }
-          base += __popc(mb);
-        }
-      }
-      __syncwarp();
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        ck[q] = lane + 32 * q < ncand ? *reinterpret_cast<const uint32_t*>(cand + q * seg + lane * 4) : 0u;
-      for (int bit = 31 - shared; bit >= 0; --bit) {
-        const uint32_t c2 = T | (1u << bit);
-        const int c = (int)__reduce_add_sync(0xffffffffu, (unsigned)((ck[0] >= c2) + (ck[1] >= c2) + (ck[2] >= c2) + (ck[3] >= c2)));
-        if (c >= m) { T = c2; if (c == m) break; }
-      }
-    } else {
-      for (int bit = 31 - shared; bit >= 0; --bit) {
-        const uint32_t c2 = T | (1u << bit);
-        const int c = count_ge(c2);
-        if (c >= m) { T = c2; if (c == m) break; }
-      }
+    for (int bit = 31 - shared; bit >= 0; --bit) {
+      const uint32_t c2 = T | (1u << bit);
+      const int c = count_ge(c2);
+      if (c >= m) { T = c2; if (c == m) break; }
     }
   }
   int base = 0, ties_seen = 0;
-  if (compacted) {
-    const uint32_t T1 = T + 1u;
-    const int need = m - (int)__reduce_add_sync(0xffffffffu, (unsigned)((ck[0] >= T1) + (ck[1] >= T1) + (ck[2] >= T1) + (ck[3] >= T1)));
+  const int need = take_all ? 0 : m - count_ge(T + 1u);
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      const bool tie = ck[q] == T, gt = ck[q] > T;
+  for (int k = 0; k < NKMAX; ++k) {
+    if (k < NK) {
+      const bool tie = !take_all && key[k] == T;
+      const bool gt = take_all ? key[k] >= kFinite : key[k] > T;
       const uint32_t mt = __ballot_sync(0xffffffffu, tie);
       const bool take = gt || (tie && ties_seen + __popc(mt & lt) < need);
       ties_seen += __popc(mt);
       const uint32_t ms = __ballot_sync(0xffffffffu, take);
-      if (take) {
-        const int j = *reinterpret_cast<const int32_t*>(cand + (4 + q) * seg + lane * 4);
-        so[base + __popc(ms & lt)] = j;
-        s[j] = -INFINITY;
-      }
+      if (take) { so[base + __popc(ms & lt)] = lane + 32 * k; s[lane + 32 * k] = -INFINITY; }
       base += __popc(ms);
-    }
-  } else {
-    const int need = take_all ? 0 : m - count_ge(T + 1u);
-#pragma unroll
-    for (int k = 0; k < NKMAX; ++k) {
-      if (k < NK) {
-        const bool tie = !take_all && key[k] == T;
-        const bool gt = take_all ? key[k] >= kFinite : key[k] > T;
-        const uint32_t mt = __ballot_sync(0xffffffffu, tie);
-        const bool take = gt || (tie && ties_seen + __popc(mt & lt) < need);
-        ties_seen += __popc(mt);
-        const uint32_t ms = __ballot_sync(0xffffffffu, take);
-        if (take) { so[base + __popc(ms & lt)] = lane + 32 * k; s[lane + 32 * k] = -INFINITY; }
-        base += __popc(ms);
-      }
     }
   }
   for (int k = base + lane; k < m; k += 32) so[k] = -1;
@@ -224,8 +283,16 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   __syncthreads();
   tc::fence_after_sync();
   const uint32_t tbase = tbase_s;
-  uint32_t cntA = 0, cntD = 0, done_ph = 0;   // tiles produced (thread 0) / consumed (thread 32) so far; phase of `done`
+  uint32_t cntA = 0, cntD = 0, done_ph = 0;   // tiles of the earlier passes (same in every thread); phase of `done`
   bool ok = true;
+  // TMA producers: lane 0 of warps 0, 2, 3, 4.  One thread sustains only about 30 bytes per clock
+  // (every bulk-tensor instruction holds it for some 270 clocks per 16 KB box, every wait after one
+  // for some 500), several threads add up.  Producer p serves the tiles whose running index is
+  // p modulo the producer count, and that count divides the ring depth, so a ring stage always
+  // belongs to one producer and its waits on the stage's barrier never fall a phase behind.
+  const int prod = lane != 0 ? -1 : warp == 0 ? 0 : (warp >= 2 && warp <= 4) ? warp - 1 : -1;
+  const int WA = nsA % 4 == 0 ? 4 : nsA % 3 == 0 ? 3 : nsA % 2 == 0 ? 2 : 1;
+  const int WD = nsD % 4 == 0 ? 4 : nsD % 2 == 0 ? 2 : 1;
   const int lq = warp & 3, tg = warp >> 2;            // TMEM lane quarter of this warp, tile group
 
   for (int r0 = p0; r0 < p1 && ok; r0 += FR) {
@@ -233,6 +300,29 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #ifdef MUSE_PHASE_CLOCKS
     long long ck0 = clock64(), ck1 = 0, ck3 = 0, ck4 = 0;
 #endif
+    // ---- A: scores^T for all clusters, kappa_hi / kappa_lo tiles through an nsA-stage TMA ring;
+    //         the producers load (TMA), thread 32 consumes (MMA), so neither waits for the other's latency.
+    //         The first ring-full of tiles is requested before the query rows are gathered.
+    // (ring stage, phase and owning producer of a tile advance by increments: no division per tile)
+    const int sA0 = cntA % nsA, phA0 = (cntA / nsA) & 1, sD0 = cntD % nsD, phD0 = (cntD / nsD) & 1;
+    int sa = sA0, pha = phA0, wa = sA0 % WA;             // of the next tile this producer looks at
+    auto next_a = [&]() {
+      if (++sa == nsA) { sa = 0; pha ^= 1; }
+      if (++wa == WA) wa = 0;
+    };
+    auto produce_a = [&](int t) {
+      const int s = sa;
+      if (!tc::mbar_wait(&bars.emptyA[s], pha ^ 1)) { ok = false; return; }
+      tc::mbar_expect_tx(&bars.fullA[s], kTileBytes);
+      const void* map = (t & 1) ? (const void*)&tm_klo : (const void*)&tm_khi;
+      const int row = (int)(ent0 + (size_t)(t >> 1) * kFJ);
+      tc::tma_load_2d(sm + s * kTileBytes, map, 0, row, &bars.fullA[s]);
+      tc::tma_load_2d(sm + s * kTileBytes + kFJ * 128, map, 64, row, &bars.fullA[s]);
+    };
+    const int TA = 2 * NJ, TA0 = min(nsA, TA);
+    if (prod >= 0 && prod < WA)
+      for (int t = 0; t < TA0 && ok; ++t, next_a())
+        if (wa == prod) produce_a(t);
     if (tid < FR) rows[tid] = tid < n ? pm[r0 + tid] : -1;
     // query rows -> K-major swizzled tile [64][128] bf16 (2 blocks of [64][128 B])
     for (int e = tid; e < FR * (kFD / 8); e += NT) {
@@ -244,48 +334,54 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     tc::fence_async_smem();
     tc::fence_before_sync();
     __syncthreads();
-    // ---- A: scores^T for all clusters, kappa_hi / kappa_lo tiles through an nsA-stage TMA ring;
-    //         thread 0 produces (TMA), thread 32 consumes (MMA), so neither waits for the other's latency
-    if (tid == 0) {
-      const int T = 2 * NJ;
-      for (int t = 0; t < T; ++t, ++cntA) {
-        const int s = cntA % nsA;
-        if (!tc::mbar_wait(&bars.emptyA[s], ((cntA / nsA) & 1) ^ 1)) { ok = false; break; }
-        tc::mbar_expect_tx(&bars.fullA[s], kTileBytes);
-        const void* map = (t & 1) ? (const void*)&tm_klo : (const void*)&tm_khi;
-        const int row = (int)(ent0 + (size_t)(t >> 1) * kFJ);
-        tc::tma_load_2d(sm + s * kTileBytes, map, 0, row, &bars.fullA[s]);
-        tc::tma_load_2d(sm + s * kTileBytes + kFJ * 128, map, 64, row, &bars.fullA[s]);
-      }
+    if (prod >= 0) {
+      if (prod < WA)
+        for (int t = TA0; t < TA && ok; ++t, next_a())
+          if (wa == prod) produce_a(t);
       // bring the nu tiles of this segment into L2 while the selection runs
-      for (int t = 0; t < NJ; ++t) {
+      for (int t = prod; t < NJ; t += 4) {
         tc::tma_prefetch_2d(&tm_nu, 0, (int)(ent0 + (size_t)t * kFJ));
         tc::tma_prefetch_2d(&tm_nu, 64, (int)(ent0 + (size_t)t * kFJ));
       }
     } else if (tid == 32) {
       tc::fence_after_sync();
       const uint32_t idesc = tc::idesc_bf16(kFJ, FR, 0, 0);
-      const uint32_t qa = tc::smem_u32(Qs);
+      const uint64_t dq0 = tc::smem_desc_sw128(tc::smem_u32(Qs), 16, 1024), da0 = tc::smem_desc_sw128(tc::smem_u32(sm), 16, 1024);
       const int T = 2 * NJ;
-      for (int u = 0; u < T; ++u, ++cntA) {
-        const int s = cntA % nsA;
-        if (!tc::mbar_wait(&bars.fullA[s], (cntA / nsA) & 1)) { ok = false; break; }
-        tc::fence_after_sync();
-        const uint32_t a0 = tc::smem_u32(sm + s * kTileBytes);
+#ifdef MUSE_PHASE_CLOCKS
+      long long ta0_ = clock64();
+#endif
+      for (int u = 0, s = sA0, ph = phA0; u < T; ++u) {
+        if (!tc::mbar_wait(&bars.fullA[s], ph)) { ok = false; break; }
+#ifdef MUSE_PHASE_CLOCKS
+        if (blockIdx.x == 200 && blockIdx.y == 5 && blockIdx.z == 1 && r0 == p0) {
+          if (u == 0) status[62] = (int)(clock64() - ta0_);
+          if (u == T - 1) status[63] = (int)(clock64() - ta0_);
+        }
+#endif
+        const uint64_t da = tc::desc_step(da0, (uint32_t)s * kTileBytes);
+        const uint32_t dcol = tbase + (u >> 1) * FR;
+
 #pragma unroll
         for (int ks = 0; ks < kFD / 16; ++ks)
-          tc::mma_bf16_ss(tbase + (u >> 1) * FR, tc::smem_desc_sw128(a0 + (ks / 4) * kFJ * 128 + (ks % 4) * 32, 16, 1024),
-                          tc::smem_desc_sw128(qa + (ks / 4) * FR * 128 + (ks % 4) * 32, 16, 1024), idesc, (u & 1) || ks > 0);
+          tc::mma_bf16_ss(dcol, tc::desc_step(da, (ks / 4) * kFJ * 128 + (ks % 4) * 32),
+                          tc::desc_step(dq0, (ks / 4) * FR * 128 + (ks % 4) * 32), idesc, (u & 1) || ks > 0);
         tc::mma_commit(&bars.emptyA[s]);
+        if (++s == nsA) { s = 0; ph ^= 1; }
       }
       if (ok) tc::mma_commit(&bars.done);
     }
     float bq[KT];                                       // beta of this thread's clusters, loaded ahead of the TMEM reads
 #pragma unroll
     for (int k = 0; k < KT; ++k) { const int jt = tg + NTG * k; bq[k] = jt < NJ ? bep[jt * kFJ + (tid & 127)] : 0.f; }
-    __syncwarp();     // lanes 1..31 of warp 0 park here instead of spinning beside the issuing lane
-    if (!tc::mbar_wait(&bars.done, done_ph)) ok = false;
+    // only the consumer polls the mbarrier; everyone else sleeps at the hardware barrier
+    if (tid == 32) {
+      if (!tc::mbar_wait(&bars.done, done_ph)) ok = false;
+      tc::fence_before_sync();
+    }
+    ok = __syncthreads_and(ok);
     done_ph ^= 1;
+    cntA += TA;
     tc::fence_after_sync();
 #ifdef MUSE_PHASE_CLOCKS
     ck1 = clock64();
@@ -325,7 +421,11 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
           for (int k = lane; k < m; k += 32) { int c = selq[k]; so[k] = c; if (c >= 0) s[c] = -INFINITY; }
         } else if (m > 0) {
           // this query's own (not yet written) P row doubles as the candidate scratch
-          select_top_m<(FR == 64 ? 32 : 64)>(s, Ck, m, so, lane, Pm + r * 128, FR * 128, Ck >= 512);
+          int* dbg = nullptr;
+#ifdef MUSE_PHASE_CLOCKS
+          if (warp == 0 && blockIdx.x == 200 && blockIdx.y == 5 && blockIdx.z == 1 && r0 == p0 && qs == 0) dbg = status + 56;
+#endif
+          select_top_m<(FR == 64 ? 32 : 64)>(s, Ck, m, so, lane, Pm + r * 128, FR * 128, Ck >= 512, dbg);
         }
         __syncwarp();
 #ifdef MUSE_PHASE_CLOCKS
@@ -356,7 +456,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       }
 #ifdef MUSE_PHASE_CLOCKS
       cb3 = clock64();
-      if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 3 && blockIdx.z == 0 && r0 == p0 && qs == 0) {
+      if (tid == 0 && blockIdx.x == 200 && blockIdx.y == 5 && blockIdx.z == 1 && r0 == p0 && qs == 0) {
         status[9] = (int)(cb1 - cb0); status[13] = (int)(cb2 - cb1); status[14] = (int)(cb3 - cb2);
       }
 #endif
@@ -369,42 +469,56 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     ck3 = clock64();
 #endif
     // ---- D: out^T = nu^T P^T, nu tiles through an nsD-stage TMA ring in the score region
-    if (tid == 0 && ok) {
+    if (prod >= 0 && prod < WD && ok) {
       unsigned char* ring = sm + p_bytes;
-      for (int t = 0; t < NJ; ++t, ++cntD) {
-        const int s = cntD % nsD;
-        if (!tc::mbar_wait(&bars.emptyD[s], ((cntD / nsD) & 1) ^ 1)) { ok = false; break; }
-        tc::mbar_expect_tx(&bars.fullD[s], kTileBytes);
+      for (int t = 0, s = sD0, ph = phD0, w = sD0 % WD; t < NJ; ++t) {
+        const int s_ = s, ph_ = ph, w_ = w;
+        if (++s == nsD) { s = 0; ph ^= 1; }
+        if (++w == WD) w = 0;
+        if (w_ != prod) continue;
+        if (!tc::mbar_wait(&bars.emptyD[s_], ph_ ^ 1)) { ok = false; break; }
+        tc::mbar_expect_tx(&bars.fullD[s_], kTileBytes);
         const int row = (int)(ent0 + (size_t)t * kFJ);
-        tc::tma_load_2d(ring + s * kTileBytes, &tm_nu, 0, row, &bars.fullD[s]);
-        tc::tma_load_2d(ring + s * kTileBytes + kFJ * 128, &tm_nu, 64, row, &bars.fullD[s]);
+        tc::tma_load_2d(ring + s_ * kTileBytes, &tm_nu, 0, row, &bars.fullD[s_]);
+        tc::tma_load_2d(ring + s_ * kTileBytes + kFJ * 128, &tm_nu, 64, row, &bars.fullD[s_]);
       }
     } else if (tid == 32 && ok) {
       tc::fence_after_sync();
       const uint32_t idesc = tc::idesc_bf16(kFD, FR, 1, 0);
-      const uint32_t pa = tc::smem_u32(Pm);
-      unsigned char* ring = sm + p_bytes;
-      for (int u = 0; u < NJ; ++u, ++cntD) {
-        const int s = cntD % nsD;
-        if (!tc::mbar_wait(&bars.fullD[s], (cntD / nsD) & 1)) { ok = false; break; }
-        tc::fence_after_sync();
-        const uint32_t a0 = tc::smem_u32(ring + s * kTileBytes);
+      const uint64_t dp0 = tc::smem_desc_sw128(tc::smem_u32(Pm), 16, 1024);
+      const uint64_t dn0 = tc::smem_desc_sw128(tc::smem_u32(sm + p_bytes), kFJ * 128, 1024);
+#ifdef MUSE_PHASE_CLOCKS
+      long long td0_ = clock64();
+#endif
+      for (int u = 0, s = sD0, ph = phD0; u < NJ; ++u) {
+        if (!tc::mbar_wait(&bars.fullD[s], ph)) { ok = false; break; }
+#ifdef MUSE_PHASE_CLOCKS
+        if (blockIdx.x == 200 && blockIdx.y == 5 && blockIdx.z == 1 && r0 == p0) {
+          if (u == 0) status[15] = (int)(clock64() - td0_);
+          if (u == NJ - 1) status[16] = (int)(clock64() - td0_);
+        }
+#endif
+        const uint64_t da = tc::desc_step(dn0, (uint32_t)s * kTileBytes), dp = tc::desc_step(dp0, (uint32_t)(2 * u) * (FR * 128));
 #pragma unroll
         for (int ks = 0; ks < kFJ / 16; ++ks)
-          tc::mma_bf16_ss(tbase, tc::smem_desc_sw128(a0 + ks * 16 * 128, kFJ * 128, 1024),
-                          tc::smem_desc_sw128(pa + (2 * u + ks / 4) * (FR * 128) + (ks % 4) * 32, 16, 1024), idesc,
+          tc::mma_bf16_ss(tbase, tc::desc_step(da, ks * 16 * 128), tc::desc_step(dp, (ks / 4) * (FR * 128) + (ks % 4) * 32), idesc,
                           u > 0 || ks > 0);
         tc::mma_commit(&bars.emptyD[s]);
+        if (++s == nsD) { s = 0; ph ^= 1; }
       }
       if (ok) tc::mma_commit(&bars.done);
     }
-    __syncwarp();
-    if (!tc::mbar_wait(&bars.done, done_ph)) ok = false;
+    if (tid == 32) {
+      if (!tc::mbar_wait(&bars.done, done_ph)) ok = false;
+      tc::fence_before_sync();
+    }
+    ok = __syncthreads_and(ok);
     done_ph ^= 1;
+    cntD += NJ;
     tc::fence_after_sync();
 #ifdef MUSE_PHASE_CLOCKS
     ck4 = clock64();
-    if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 3 && blockIdx.z == 0 && r0 == p0) {
+    if (tid == 0 && blockIdx.x == 200 && blockIdx.y == 5 && blockIdx.z == 1 && r0 == p0) {
       status[8] = (int)(ck1 - ck0); status[9] = 0; status[10] = (int)(ck3 - ck1); status[11] = (int)(ck4 - ck3);
       status[12] = n;
     }
