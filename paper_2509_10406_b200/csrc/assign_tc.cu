@@ -64,38 +64,39 @@ k_assign_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
     if (tid == 8 * 32) {                                   // ---- producer
       tc::mbar_expect_tx(&bars.xbar, kX);
       for (int g = 0; g < D / 64; ++g) tc::tma_load_2d(Xs + g * kAtRows * 128, &tm_x, 64 * g, prob * N + row0, &bars.xbar);
-      for (int t = 0; t < NT && ok; ++t) {
-        const int s = t % ns;
-        if (!tc::mbar_wait(&bars.empty[s], ((t / ns) & 1) ^ 1)) { ok = false; break; }
+      for (int t = 0, s = 0, ph = 0; t < NT && ok; ++t) {                // (stage and phase by increments: no division per tile)
+        if (!tc::mbar_wait(&bars.empty[s], ph ^ 1)) { ok = false; break; }
         tc::mbar_expect_tx(&bars.full[s], kStage);
         unsigned char* st = ring + s * kStage;
         for (int g = 0; g < D / 64; ++g) {
           tc::tma_load_2d(st + g * kAtCols * 128, &tm_hi, 64 * g, prob * C + t * kAtCols, &bars.full[s]);
           tc::tma_load_2d(st + kC + g * kAtCols * 128, &tm_lo, 64 * g, prob * C + t * kAtCols, &bars.full[s]);
         }
+        if (++s == ns) { s = 0; ph ^= 1; }
       }
     }
   } else if (warp == 9) {
     if (tid == 9 * 32) {                                   // ---- MMA issuer
       const uint32_t idesc = tc::idesc_bf16(kAtRows, kAtCols, 0, 0);
-      const uint32_t xa = tc::smem_u32(Xs);
+      const uint64_t dx0 = tc::smem_desc_sw128(tc::smem_u32(Xs), 16, 1024), dr0 = tc::smem_desc_sw128(tc::smem_u32(ring), 16, 1024);
       if (!tc::mbar_wait(&bars.xbar, 0)) ok = false;
-      for (int t = 0; t < NT && ok; ++t) {
-        const int s = t % ns, b = t & 1;
+      for (int t = 0, s = 0, ph = 0; t < NT && ok; ++t) {
+        const int b = t & 1;
         if (!tc::mbar_wait(&bars.tempty[b], ((t >> 1) & 1) ^ 1)) { ok = false; break; }
-        if (!tc::mbar_wait(&bars.full[s], (t / ns) & 1)) { ok = false; break; }
+        if (!tc::mbar_wait(&bars.full[s], ph)) { ok = false; break; }
         tc::fence_after_sync();
-        const uint32_t ha = tc::smem_u32(ring + s * kStage), la = ha + kC;
+        const uint64_t dh = tc::desc_step(dr0, (uint32_t)s * kStage), dl = tc::desc_step(dh, kC);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks)
-          tc::mma_bf16_ss(tbase + b * kAtCols, tc::smem_desc_sw128(xa + (ks / 4) * kAtRows * 128 + (ks % 4) * 32, 16, 1024),
-                          tc::smem_desc_sw128(ha + (ks / 4) * kAtCols * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
+          tc::mma_bf16_ss(tbase + b * kAtCols, tc::desc_step(dx0, (ks / 4) * kAtRows * 128 + (ks % 4) * 32),
+                          tc::desc_step(dh, (ks / 4) * kAtCols * 128 + (ks % 4) * 32), idesc, ks > 0);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks)
-          tc::mma_bf16_ss(tbase + b * kAtCols, tc::smem_desc_sw128(xa + (ks / 4) * kAtRows * 128 + (ks % 4) * 32, 16, 1024),
-                          tc::smem_desc_sw128(la + (ks / 4) * kAtCols * 128 + (ks % 4) * 32, 16, 1024), idesc, 1);
+          tc::mma_bf16_ss(tbase + b * kAtCols, tc::desc_step(dx0, (ks / 4) * kAtRows * 128 + (ks % 4) * 32),
+                          tc::desc_step(dl, (ks / 4) * kAtCols * 128 + (ks % 4) * 32), idesc, 1);
         tc::mma_commit(&bars.empty[s]);                    // the centre tiles may be overwritten ...
         tc::mma_commit(&bars.tfull[b]);                    // ... and the distances read
+        if (++s == ns) { s = 0; ph ^= 1; }
       }
     }
   } else {
