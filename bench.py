@@ -221,9 +221,9 @@ def workload_config(w, gain):
 # DRAM bytes per (batch, head) problem from the ncu capture of the headline workload cut to one
 # head (dram__bytes_read.sum + dram__bytes_write.sum; the capture's command and figures are in
 # profiles/top_kernels_headline_one_head.md).  Traffic grows in proportion to the problem count.
-NCU_TRAFFIC_PER_HEAD = {"k_summarize_tc": 1.432e9, "k_local_fwd_tc": 0.054e9, "k_far_fwd_tc": 1.682e9,
-                        "k_ret_bwd_fused_tc": 0.610e9, "k_ret_fwd_cluster_tc": 0.524e9, "k_far_bwd_tc": 2.412e9,
-                        "k_summ_bwd_tc": 1.102e9, "k_local_bwd_dkdv_tc": 0.090e9, "k_local_bwd_dq_tc": 0.073e9}
+NCU_TRAFFIC_PER_HEAD = {"k_summarize_tc": 1.430e9, "k_local_fwd_tc": 0.056e9, "k_far_fwd_tc": 1.634e9,
+                        "k_ret_bwd_fused_tc": 0.608e9, "k_ret_fwd_cluster_tc": 0.529e9, "k_far_bwd_tc": 2.411e9,
+                        "k_summ_bwd_tc": 1.102e9, "k_local_bwd_dkdv_tc": 0.088e9, "k_local_bwd_dq_tc": 0.073e9}
 
 
 def main():
