@@ -220,7 +220,9 @@ k_local_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_k, const __grid_c
   const uint32_t tbase = tbase_s, tl = tbase + ((uint32_t)((warp & 3) * 32) << 16);
   const uint32_t qa = tc::smem_u32(Qs), ka = tc::smem_u32(Ks), va = tc::smem_u32(Vs), pa = tc::smem_u32(Ps);
   bool ok = true;
-  // thread 0 only: tile loads and MMA issue.  Rows past the block's visible keys are loaded too (they are masked).
+  // Thread 0 issues the MMAs, thread 32 the tile loads: a bulk-tensor instruction holds its thread for some
+  // 270 clocks per 16 KB box, and every row of the tile waits for thread 0 at the next barrier.
+  // Rows past the block's visible keys are loaded too (they are masked).
   auto load_k = [&](int t) {
     tc::mbar_expect_tx(&barK[t & 1], kKB);
     for (int g = 0; g < D / 64; ++g) tc::tma_load_2d(Ks + (t & 1) * kKB + g * kTcN * 128, &tm_k, 64 * g, krow0 + t * kTcN, &barK[t & 1]);
@@ -240,11 +242,11 @@ k_local_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_k, const __grid_c
                       tc::smem_desc_sw128(kat + (ks / 4) * kTcN * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
     tc::mma_commit(&barS[t & 1]);
   };
-  if (tid == 0) {
+  if (tid == 32) {
     load_k(0);
     if (T > 1) load_k(1);
-    issue_s(0);
   }
+  if (tid == 0) issue_s(0);
   const float scale2 = dm.sigma * 1.4426950408889634f;
   const int my_limit = q0 + row;                            // last visible key of this row
   // The output accumulates in TMEM over all key tiles.  m2 is the exponent base in use for this row (log2
@@ -262,7 +264,7 @@ k_local_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_k, const __grid_c
       if (!tc::mbar_wait(&barPV, (t - 1) & 1)) ok = false;
       tc::fence_after_sync();
     }
-    if (tid == 0) {
+    if (tid == 32) {
       load_v(t);
       if (t + 2 < T) load_k(t + 2);                         // over K_t, which S(t) has consumed
     }
