@@ -135,3 +135,33 @@ def test_forward_per_query_cluster_selection():
 
 def test_forward_noncausal():
     _forward_parity(CASES["tiny"], 128.0, causal=False)
+
+
+@pytest.mark.parametrize("groups", [8, 2])
+def test_selection_with_exact_ties_takes_the_lowest_cluster_indices(groups):
+    """Key clusters with identical contents have bit-identical summaries and scores, on both sides.  512
+    clusters in `groups` classes: the threshold of the top 32 falls inside a class of 64 (compacted selection,
+    more ties than places) or 256 (too many candidates to compact: the general path).  Both sides break ties
+    towards the lowest cluster index, so the selected sets must be equal for every query."""
+    w = CASES["d128"].with_(Hq=1, Hkv=1, N=8192, S=4, Cq=8, Ck=512, m=32)
+    mb, c, p, buf = _prep(w, 128.0)
+    rng = np.random.default_rng(1234 + groups)
+    t = np.arange(w.N)
+    bf = lambda x: to_np(torch.from_numpy(x.astype(np.float32)).to(torch.bfloat16)).astype(np.float32)
+    proto_k = bf(rng.standard_normal((w.N // w.Ck, groups, w.D)) * 2.0)       # [round][class][D]
+    proto_v = bf(rng.standard_normal((w.N // w.Ck, groups, w.D)))
+    c.K[0, 0] = proto_k[t // w.Ck, (t % w.Ck) % groups]
+    c.V[0, 0] = proto_v[t // w.Ck, (t % w.Ck) % groups]
+    c.a_k[0, 0] = (t % w.Ck).astype(np.int32)
+    Q, K, V, _ = c.dev()
+    _run_summaries(mb, c, p, buf, K, V)
+    mb.muse_attn_fwd(p, Q, K, V, to_dev(c.a_q, "i"), to_dev(c.qbar32, "f32"), buf.off_k, buf.perm_k, buf.summaries,
+                     None, buf.O, buf.LSE, buf.sel, buf.ws)
+    torch.cuda.synchronize()
+    sel_gpu = to_np(buf.sel)[0, 0, :, :w.m]
+    f = orc.forward(c.Q[0, 0], c.K[0, 0], c.V[0, 0], c.a_q[0, 0], c.a_k[0, 0], c.qbar32[0, 0].astype(np.float64),
+                    sigma=c.sigma, S=w.S, Ck=w.Ck, m=w.m)
+    rows = np.arange(w.N // w.S, w.N)                    # the first block has no far field
+    differ = [r for r in rows if set(sel_gpu[r].tolist()) != set(f["sel"][r].tolist())]
+    assert not differ, (len(differ), differ[:5], sorted(sel_gpu[differ[0]].tolist()), sorted(f["sel"][differ[0]].tolist()))
+    assert rel_err(to_np(buf.O)[0, 0], f["O"]) <= tol(w.dtype)
