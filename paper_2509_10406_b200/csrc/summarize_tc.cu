@@ -91,7 +91,7 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
 #endif
 
   // The cluster's keys are contiguous in bucket order, so its chunks (at most 64 keys, never across a
-  // bucket boundary) form one sequence; thread 0 starts the load of chunk n + 1 as soon as the MMAs of
+  // bucket boundary) form one sequence; thread 32 starts the load of chunk n + 1 as soon as the MMAs of
   // chunk n have released the key / value tiles, so that it lands while the snapshot is written.
   // A bucket usually holds far fewer than 64 keys: only the 16-key groups in use are loaded and contracted.
   auto issue_kv = [&](int c0, int nk) {
@@ -108,7 +108,7 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
     while (npl < dm.SB && off[npl + 1] <= c_end) ++npl;
     if (npl < dm.SB) issue_kv(c_end, min(NU, off[npl + 1] - c_end));
   };
-  if (tid == 0) issue_after(off[0]);
+  if (tid == 32) issue_after(off[0]);
   for (int pl = 0; pl < dm.SB && ok; ++pl) {
     const int p0 = off[pl], p1 = off[pl + 1];
     for (int c0 = p0; c0 < p1 && ok; c0 += NU) {
@@ -188,7 +188,7 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
       if (!tc::mbar_wait(&bar2, ph2)) ok = false;
       ph2 ^= 1;
       tc::fence_after_sync();
-      if (tid == 0 && ok) issue_after(c0 + nk);          // key / value tiles are free again
+      if (tid == 32 && ok) issue_after(c0 + nk);         // key / value tiles are free again (not thread 0: it issues the MMAs)
       PCLK(3)
 #pragma unroll
       for (int d0 = 0; d0 < D; d0 += 32) {              // acc[0..63]: kappa dims 64 wg.., acc[64..127]: nu dims 64 wg..
