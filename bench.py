@@ -42,9 +42,11 @@ def work_model(w: wl.Workload):
     nd = N * D
     ret_keys = m * (N / Ck) * (S - 1) / (2 * S)             # nominal retrieved keys per query
     local = 2 * D * N * Bs                                  # 2 matmuls over the causal half
-    far_tc = w.dtype == "bf16" and D == 128 and Ck % 128 == 0 and Ck <= 2048      # tensor-core far-field path
-    summ = heads * SB * Cq * Ck * ((3 * D * 2 + 8) if far_tc else (2 * D + 1) * 4)  # accumulated summaries
-    grads = heads * SB * Cq * Ck * ((2 * D * 2 + 4) if far_tc else (2 * D + 1) * 4) # their gradients
+    # Accumulated summaries as the method defines them: (mu, kappa[D], nu[D]) per (head, plane, i, j) in the
+    # storage type e' (bf16 / fp32); their gradients have the same shape.  What the kernels move on top of
+    # that (a second kappa plane, beta) is implementation traffic: see impl_bytes().
+    summ = heads * SB * Cq * Ck * (2 * D + 1) * e
+    grads = heads * SB * Cq * Ck * (2 * D + 1) * e
     part = heads * N * m * D * (2 if w.dtype == "bf16" else 4)                       # retrieval partials (o or dq)
     M = {
         # clustering
@@ -88,6 +90,32 @@ def work_model(w: wl.Workload):
         "k_dipole_apply": ("hbm", heads * SB * Cq * D * D * e + heads * nd * (e + 8)),
     }
     return M
+
+
+def impl_bytes(w: wl.Workload):
+    """Bytes the summary-streaming kernels actually move per step in this implementation (stored layout),
+    for comparison with the algorithmic bytes of work_model: the difference is overhead, not work."""
+    B, Hq, Hkv, N, D, Cq, Ck, S = w.B, w.Hq, w.Hkv, w.N, w.D, w.Cq, w.Ck, w.S
+    e = 4 if w.dtype == "f32" else 2
+    heads, kvh, nd, ent = B * Hq, B * Hkv, N * D, B * Hq * (S - 1) * Cq * Ck
+    st = stored_summary_bytes_per_entry(w)
+    gr = (2 * D * 2 + 4) if w.dtype == "bf16" else (2 * D + 1) * 4
+    return {"k_summarize_tc": ent * st + 2 * kvh * nd * e, "k_summarize": ent * st + 2 * kvh * nd * e,
+            "k_far_fwd_tc": ent * st + heads * nd * (e + 4), "k_far_fwd": ent * st + heads * nd * (e + 4),
+            "k_far_bwd_tc": ent * (st + gr) + heads * nd * (2 * e + 8), "k_far_bwd": ent * (st + gr) + heads * nd * (2 * e + 8),
+            "k_summ_bwd_tc": ent * gr + 2 * kvh * nd * e + 4 * heads * nd * 4, "k_summ_bwd": ent * gr + 2 * kvh * nd * e + 4 * heads * nd * 4}
+
+
+def stored_summary_bytes_per_entry(w: wl.Workload) -> int:
+    if w.dtype == "f32":
+        return (2 * w.D + 2) * 4
+    return SUMMARY_KAPPA_PLANES * w.D * 2 + w.D * 2 + 8       # kappa plane(s) + nu, bf16; mu and beta fp32
+
+
+SUMMARY_KAPPA_PLANES = 2      # bf16 mode stores kappa as a hi + lo pair
+
+
+NOMINAL = dict(hbm=8000.0, tensor=2250.0)     # "roughly 8 TB/s" and the dense bf16 peak, for context
 
 
 def peaks():
@@ -157,21 +185,46 @@ def gen_inputs(w: wl.Workload, gain: float):
     return Q, K, V, dO, iq, ik
 
 
-def oracle_sample_seconds(w: wl.Workload, gain: float, rows_n: int):
+def oracle_sample_seconds(w: wl.Workload, gain: float, rows_n: int, gpu=None):
     """Times the fp64 oracle, as it stands, on one (batch 0, head 0) problem: full clustering and
     summaries, forward+backward for `rows_n` sampled queries; scales the per-query part to N
-    queries and everything to all heads.  Returns (estimated seconds per step, description)."""
+    queries and everything to all heads.  Returns (estimated seconds per step, description, stats).
+    `gpu` (optional): the CUDA path's results for that head (assign_q, assign_k, qbar, kcent, sel, O, dQ as
+    numpy arrays).  The oracle's per-query part then runs on the GPU's clustering, so that its selections
+    and outputs for the sampled queries can be compared with the GPU's (reported statistics, not a gate)."""
     from oracle import muse_oracle as orc
     Q, K, V, dO = (x.astype(np.float64) for x in wl.make_head_inputs(w, 0, 0, gain=gain))
     iq = wl.random_init_indices(w.N, w.Cq, w.seed, 0); ik = wl.random_init_indices(w.N, w.Ck, w.seed, 1)
     sigma = 1.0 / np.sqrt(w.D)
     t0 = time.perf_counter()
     a_q, qbar = orc.lloyd(Q, w.T, init_idx=iq)
-    a_k, _ = orc.lloyd(K, w.T, init_idx=ik)
+    a_k, kcent = orc.lloyd(K, w.T, init_idx=ik)
     t1 = time.perf_counter()
     rows = np.sort(np.random.default_rng(0).choice(w.N, size=min(rows_n, w.N), replace=False))
-    dQ, dK, dV, _ = orc.backward(Q, K, V, dO, a_q, a_k, qbar, sigma=sigma, S=w.S, Ck=w.Ck, m=w.m, rows=rows)
+    stats = None
+    if gpu is not None:
+        stats = {"free_running_lloyd_assignments_differing": int((gpu["assign_q"] != a_q).sum() + (gpu["assign_k"] != a_k).sum()),
+                 "of": int(a_q.size + a_k.size)}
+        pts = np.sort(np.random.default_rng(1).choice(w.N, size=min(4096, w.N), replace=False))
+        near = bad = 0
+        for X, a, c in ((Q, gpu["assign_q"], gpu["qbar"]), (K, gpu["assign_k"], gpu["kcent"])):
+            gaps = orc.assignment_gaps(X[pts], c.astype(np.float64))
+            near += int((gaps < 1e-4).sum())
+            bad += int((orc.assign_nearest(X[pts], c.astype(np.float64)) != a[pts]).sum())
+        stats.update(sampled_points=int(2 * pts.size), near_tie_assignments=near, assignments_differing_from_fp64_argmin=bad)
+        a_q, a_k, qbar = gpu["assign_q"], gpu["assign_k"], gpu["qbar"].astype(np.float64)
+    dQ, dK, dV, f = orc.backward(Q, K, V, dO, a_q, a_k, qbar, sigma=sigma, S=w.S, Ck=w.Ck, m=w.m, rows=rows)
     t2 = time.perf_counter()
+    if gpu is not None and w.m > 0:
+        same = np.array([set(f["sel"][t].tolist()) == set(gpu["sel"][t].tolist()) for t in rows])
+        gap = f["sel_gap"][rows][~same]
+        stats.update(sampled_queries=int(rows.size), selection_rows_differing=int((~same).sum()),
+                     largest_oracle_margin_where_differing=float(gap.max()) if gap.size else 0.0)
+        ok_rows = rows[same]
+        if ok_rows.size:
+            rel = lambda x, r: float(np.abs(x - r).max() / max(np.abs(r).max(), 1e-30))
+            stats.update(O_err_rows_with_equal_selection=rel(gpu["O"][ok_rows], f["O"][ok_rows]),
+                         dQ_err_rows_with_equal_selection=rel(gpu["dQ"][ok_rows], dQ[ok_rows]) if gpu.get("dQ") is not None else None)
     # backward() = summaries + per-query forward/backward of the sampled rows + key-side pass;
     # time the row-independent part separately to scale only the per-query part
     t3 = time.perf_counter()
@@ -183,7 +236,7 @@ def oracle_sample_seconds(w: wl.Workload, gain: float, rows_n: int):
     desc = (f"batch 0 / head 0 of '{w.name}': Lloyd T={w.T} on Q and K ({t1 - t0:.1f}s), summaries + key-side "
             f"backward ({fixed:.1f}s), forward+backward of {len(rows)} sampled queries ({per_row * 1e3:.1f} ms/query); "
             f"per-query part scaled to N={w.N}, all scaled to {w.B * w.Hq} heads")
-    return est, desc
+    return est, desc, stats
 
 
 def run_reference(args, w, gain):
@@ -195,7 +248,7 @@ def run_reference(args, w, gain):
     cores = torch.get_num_threads()
     times = []
     for k in range(args.warmup + args.steps):
-        est, desc = oracle_sample_seconds(w, gain, args.ref_rows)
+        est, desc, _ = oracle_sample_seconds(w, gain, args.ref_rows)
         if k >= args.warmup:
             times.append(est)
     t = statistics.mean(times)
@@ -218,9 +271,9 @@ def workload_config(w, gain):
             "parallelism": "replicas"}
 
 
-# DRAM bytes per (batch, head) problem from the ncu capture of the headline workload cut to one
-# head (dram__bytes_read.sum + dram__bytes_write.sum; the capture's command and figures are in
-# profiles/top_kernels_headline_one_head.md).  Traffic grows in proportion to the problem count.
+# DRAM bytes per (batch, head) problem from an ncu capture (--set full) of the headline workload cut
+# to one head: dram__bytes_read.sum + dram__bytes_write.sum per launch.  Traffic grows in proportion
+# to the problem count.
 NCU_TRAFFIC_PER_HEAD = {"k_summarize_tc": 1.430e9, "k_local_fwd_tc": 0.056e9, "k_far_fwd_tc": 1.634e9,
                         "k_ret_bwd_fused_tc": 0.608e9, "k_ret_fwd_cluster_tc": 0.529e9, "k_far_bwd_tc": 2.411e9,
                         "k_summ_bwd_tc": 1.102e9, "k_local_bwd_dkdv_tc": 0.088e9, "k_local_bwd_dq_tc": 0.073e9}
@@ -247,6 +300,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sharp", action="store_true", help="skip the extra timing on the sharp variant of the inputs")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "muse" else args.warmup
 
@@ -364,6 +418,15 @@ def main():
         ms = float(t.item())
     tokens = w.B * w.N
     value = world * tokens / (ms * 1e-3)
+    O_first = O_all.clone() if (groups == 1 and not args.no_dense) else None
+    dev_status = mb.muse_status(buf.ws)           # 0 = no kernel of the last call reported a wait that ran out
+    # the CUDA path's results for (batch 0, head 0), for the reported parity statistics
+    gpu_head0 = None
+    if rank == 0 and groups == 1 and not args.no_cpu_baseline:
+        npy = lambda t: t.detach().float().cpu().numpy() if t.dtype in (torch.bfloat16, torch.float32) else t.cpu().numpy()
+        gpu_head0 = dict(assign_q=npy(buf.assign_q[0, 0]), assign_k=npy(buf.assign_k[0, 0]), qbar=npy(buf.qbar[0, 0]),
+                         kcent=npy(buf.kcent[0, 0]), sel=npy(buf.sel[0, 0])[:, :max(w.m, 0)], O=npy(O_all[0, 0]),
+                         dQ=None if args.forward_only else npy(dQ_all[0, 0]))
 
     # end to end: host buffers in, host buffers out, through the same public calls
     e2e = None
@@ -449,8 +512,7 @@ def main():
         e2e = {"value": world * tokens / (ems * 1e-3), "unit": UNIT, "ms_per_step": ems,
                "h2d_bytes_per_step": nb(hQ, hK, hV, hdO), "d2h_bytes_per_step": nb(*[h for h, _ in outs]),
                "head_stages": eg, "copy_streams": 2,
-               # (not bit-equal in general: the centroid update adds with floating-point atomics, so two runs
-               # can differ in near-tie assignments)
+               # (the two runs pass different numbers of heads per call)
                "output_max_abs_diff_vs_device_run_rel": float(((hO.cuda().float() - O_dev.float()).abs().max()
                                                                 / O_dev.float().abs().max()).item())}
         del O_dev
@@ -481,7 +543,9 @@ def main():
             traffic = NCU_TRAFFIC_PER_HEAD[top] * w.B * w.Hq    # one launch per step covers all heads
         roof.update(bound=bound, achieved=ach, peak=peak, unit=unit, frac=ach / peak, traffic=traffic,
                     peak_source=pk["source"] + (" (sustained bf16)" if bound == "tensor" else " (copy)"),
+                    frac_of_nominal=ach / NOMINAL[bound], nominal_peak=NOMINAL[bound],
                     algorithmic_work_per_step=work, kernel_ms_per_step=kernels[top]["ms_per_step"])
+    impl = impl_bytes(w)
     for k, v in kernels.items():
         if k in model:
             bound, work = model[k]
@@ -489,6 +553,10 @@ def main():
             v["bound"] = bound
             v["achieved"] = work / sec / (1e12 if bound == "tensor" else 1e9)
             v["frac"] = v["achieved"] / (pk["tensor_sustained"] if bound == "tensor" else pk["hbm"])
+            v["frac_of_nominal"] = v["achieved"] / NOMINAL[bound]
+            if k in impl:                        # bytes the stored layout makes the kernel move, beside the algorithmic ones
+                v["implementation_gbs"] = impl[k] / sec / 1e9
+                v["implementation_over_algorithmic_bytes"] = impl[k] / work
 
     context = {}
     if not args.no_dense:
@@ -502,23 +570,68 @@ def main():
                 o = F.scaled_dot_product_attention(q, k, v, is_causal=True)
                 o.backward(dO)
                 q.grad = k.grad = v.grad = None
+                return o
             dense(); torch.cuda.synchronize()
             ev0.record()
             for _ in range(3):
-                dense()
+                o_dense = dense()
             ev1.record(); torch.cuda.synchronize()
             dms = ev0.elapsed_time(ev1) / 3
             context["dense_sdpa_fwd_bwd_ms"] = dms
             context["speedup_vs_dense_sdpa"] = dms / ms
-            del q, k, v
+            if groups == 1 and O_first is not None:
+                # relative squared error of the approximation against exact attention, averaged over queries
+                # (Appendix "Hyperparameters", "Evaluation metrics"); context only: synthetic mixtures have none of
+                # the structure of trained-model attention
+                od = o_dense.detach().float()
+                num = (O_first.float() - od).pow(2).sum(-1); den = od.pow(2).sum(-1).clamp_min(1e-30)
+                context["rse_vs_dense_mean_over_queries"] = float((num / den).mean().item())
+            del q, k, v, o_dense
         except Exception as ex:  # bench-only comparator; never fatal
             context["dense_sdpa_error"] = repr(ex)[:200]
+        try:
+            # exact causal attention through this library's own kernels: one spatial block, nothing retrieved,
+            # no far field (the block-diagonal kernels then cover the whole sequence)
+            pd = mb.make_params(B=w.B, Hq=w.Hq, Hkv=w.Hkv, N=w.N, D=w.D, Cq=1, Ck=1, m=0, n_blocks=1, dtype=w.dtype,
+                                kmeans_iters=0, init_mode=mb.MUSE_INIT_STRIDED)
+            bd = mb.MuseBuffers(pd, backward=True)
+            mb.muse_cluster(pd, Q, K, None, None, bd.assign_q, bd.assign_k, bd.qbar, bd.kcent, bd.ws)
+            mb.muse_summarize(pd, K, V, bd.assign_k, bd.qbar, bd.off_k, bd.perm_k, bd.summaries, bd.ws)
+
+            def own():
+                mb.muse_attn_fwd(pd, Q, K, V, bd.assign_q, bd.qbar, bd.off_k, bd.perm_k, bd.summaries, None, bd.O, bd.LSE, bd.sel, bd.ws)
+                mb.muse_attn_bwd(pd, Q, K, V, bd.O, bd.LSE, dO, bd.assign_q, bd.qbar, bd.off_k, bd.perm_k, bd.summaries, bd.sel,
+                                 bd.dQ, bd.dK, bd.dV, bd.ws)
+            own(); torch.cuda.synchronize()
+            ev0.record()
+            for _ in range(3):
+                own()
+            ev1.record(); torch.cuda.synchronize()
+            context["dense_own_kernels_fwd_bwd_ms"] = ev0.elapsed_time(ev1) / 3
+            del bd
+        except Exception as ex:
+            context["dense_own_kernels_error"] = repr(ex)[:200]
+    if not args.no_sharp and args.gain == 1.0:
+        # the same step on the sharp variant of the inputs (Q x 128, exact in bf16): attention is then peaked,
+        # so selection and retrieval matter; k-means and the tile schedule are scale-free
+        Q.mul_(128.0)
+        for _ in range(2):
+            step()
+        torch.cuda.synchronize()
+        ev0.record()
+        for _ in range(3):
+            step()
+        ev1.record(); torch.cuda.synchronize()
+        context["sharp_inputs_ms_per_step"] = ev0.elapsed_time(ev1) / 3
+        context["sharp_inputs_device_status"] = mb.muse_status(buf.ws)
+        Q.mul_(1.0 / 128.0)
     context["paper"] = ("2x over cuDNN flash attention at 64k and +36% pretraining throughput, 8xA100, "
                         "D=64, QK128R8SP1B8k (other hardware and configuration: context only)")
 
     cpu = None
+    parity_stats = None
     if not args.no_cpu_baseline:
-        est, desc = oracle_sample_seconds(w, args.gain, args.ref_rows)
+        est, desc, parity_stats = oracle_sample_seconds(w, args.gain, args.ref_rows, gpu=gpu_head0)
         cpu = {"value": tokens / est, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                "sample": desc, "est_seconds_per_step": est}
 
@@ -529,7 +642,8 @@ def main():
                            dipole=int(args.dipole), passes="cluster+summarize+forward" if args.forward_only else "cluster+summarize+forward+backward"),
             "ms_per_step_median": statistics.median(per_step), "ms_per_step_best": min(per_step), "stages_ms": stages,
             "clocks": clocks, "e2e": e2e,
-            "gpu_launches": launches, "roofline": roof, "cpu_baseline": cpu, "kernels": kernels, "context": context}
+            "gpu_launches": launches, "roofline": roof, "cpu_baseline": cpu, "kernels": kernels, "context": context,
+            "device_status": dev_status, "parity_stats_head0": parity_stats}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -24,6 +24,17 @@
  *     calls on the same stream.  Pointers must be 16-byte aligned.
  *   - Return value: MUSE_OK (0) or a negative MUSE_ERR_* code.  Arguments are checked on the
  *     host before anything is launched; nothing aborts or throws.
+ *   - Device status.  Inside the kernels every wait on the hardware (a tensor-core or copy
+ *     completion barrier) is bounded by elapsed SM clocks (about half a second); a wait that runs out
+ *     makes its kernel stop early instead of hanging the GPU, and the outputs of that call are then
+ *     undefined.  The first 64 int32 words of `ws` are status words: each entry point clears them
+ *     when it starts, word 0 receives the first MUSE_STATUS_* code a kernel of the call reported
+ *     (0 = the call ran to completion), the other words are reserved.  The word is written
+ *     asynchronously: read it after synchronising the stream, directly from `ws` or through
+ *     muse_status_copy.  Indices supplied by the caller are never trusted as addresses: an
+ *     assignment outside [0, C) is treated as the nearest valid cluster index and a selection entry
+ *     outside [0, Ck) as -1 (none); a row of Q or K that holds NaN or infinities is assigned to
+ *     cluster 0.
  *   - Spatial blocks: block(t) = t / (N / n_blocks).  Keys are bucketed cluster-major,
  *     block-minor: bucket (j,b) occupies positions [off_k[j*S+b], off_k[j*S+b+1]) of the
  *     permutation perm_k (position -> original key index, stable, i.e. ascending inside a
@@ -52,6 +63,18 @@ typedef struct CUstream_st* cudaStream_t;
 enum { MUSE_BF16 = 0, MUSE_F32 = 1 };
 enum { MUSE_SEL_PER_QUERY = 0, MUSE_SEL_PER_QCLUSTER = 1 };
 enum { MUSE_INIT_INDICES = 0, MUSE_INIT_STRIDED = 1, MUSE_INIT_CENTRES = 2 };
+/* Device status word (see "Device status" below): first code reported by a kernel of the call. */
+enum {
+  MUSE_STATUS_OK = 0,
+  MUSE_STATUS_FWD_TIMEOUT = 1,       /* exact-attention forward kernels (local, retrieval)         */
+  MUSE_STATUS_BWD_TIMEOUT = 2,       /* exact-attention backward kernels                           */
+  MUSE_STATUS_FAR_FWD_TIMEOUT = 3,   /* far-field forward (scores, top-m, approximate attention)   */
+  MUSE_STATUS_FAR_BWD_TIMEOUT = 4,   /* far-field backward                                         */
+  MUSE_STATUS_SUMM_BWD_TIMEOUT = 5,  /* key-side pass through the summaries                        */
+  MUSE_STATUS_ASSIGN_TIMEOUT = 6,    /* k-means assignment                                         */
+  MUSE_STATUS_SUMM_TIMEOUT = 7,      /* summaries / dipole construction                            */
+  MUSE_STATUS_SELFTEST_TIMEOUT = 9   /* muse_test_wait_timeout                                     */
+};
 enum {
   MUSE_OK = 0,
   MUSE_ERR_INVALID_ARG = -1,   /* null pointer, bad size, misaligned pointer            */
@@ -81,11 +104,12 @@ typedef struct muse_params {
 } muse_params_t;
 
 /* Sizes in bytes of the scratch each stage needs and of the opaque summaries buffer.
- * out[0] cluster, out[1] summarize, out[2] attn_fwd, out[3] attn_bwd, out[4] summaries.
+ * out[0] cluster, out[1] summarize, out[2] attn_fwd, out[3] attn_bwd, out[4] summaries,
+ * out[5] attn_bwd when it is called with summaries == NULL and rebuilds them in its scratch.
  * Appendix "Clustering Cost" / Section "Summary Computation": the summaries buffer holds the
  * S-1 accumulated (mu, beta, kappa, nu) planes over [B,Hq,S-1,Cq,Ck], followed by the bucketed
  * copies of K and V (see muse_summaries_layout). */
-MUSE_API int muse_workspace_bytes(const muse_params_t* p, size_t out[5]);
+MUSE_API int muse_workspace_bytes(const muse_params_t* p, size_t out[6]);
 
 /* Byte offsets inside the summaries buffer, per entry e = (b, h, plane, i, j) of
  * [B,Hq,SB,Cq,Ck], SB = S-1 (causal) or 1; plane s is the accumulated summary seen by queries
@@ -120,16 +144,20 @@ MUSE_API int muse_cluster(const muse_params_t* p, const void* Q, const void* K,
 
 /* Clustering without a caller-provided workspace (the paper has no counterpart; this is a
  * deployment aid).  Same inputs, outputs and results as muse_cluster, but the scratch memory is
- * a fixed 32 MiB array built into the library's device image, so the call performs no device
- * allocation of any kind and needs no scratch pointer.  It is meant for callers that cannot
+ * a fixed 32 MiB array built into the library's device image, so the call itself makes no
+ * allocation request of any kind and needs no scratch pointer.  It is meant for callers that cannot
  * allocate or own no spare device memory: code running inside a serving loop where a device
  * allocation would stall every stream, plugins living under a framework whose pool already
  * owns the whole GPU, or hosts that must not fail with out-of-memory in mid-request.
  *   - Every GPU that loads the library carries the 32 MiB until the process exits.
  *   - Problems whose clustering scratch (muse_workspace_bytes out[0]) exceeds
  *     muse_cluster_noalloc_max_bytes() are rejected with MUSE_ERR_WORKSPACE; nothing is launched.
- *   - The first call on each device looks up the array's device address (the device must be
- *     current); make that first call outside any stream capture.
+ *   - Every call looks up the array's device address for the current device.  The first lookup on
+ *     a device loads the library's device image there, and that is when the driver reserves the
+ *     32 MiB: this first call can therefore return MUSE_ERR_CUDA (no memory left for the image) and
+ *     should be made before any stream capture.  Later calls only read a host-side table.
+ *   - The status word of the call sits inside the built-in array: muse_cluster_noalloc_status_copy
+ *     enqueues its copy to memory the caller owns.
  *   - All calls share the one array and find in it whatever the previous call left; the stage
  *     clears what it needs zeroed itself.  Two calls that overlap on the GPU (different streams,
  *     or different threads) race on it: serialise them. */
@@ -138,6 +166,11 @@ MUSE_API int muse_cluster_noalloc(const muse_params_t* p, const void* Q, const v
                          int32_t* assign_q, int32_t* assign_k, float* qbar, float* kcent,
                          cudaStream_t stream);
 MUSE_API size_t muse_cluster_noalloc_max_bytes(void);
+MUSE_API int muse_cluster_noalloc_status_copy(int32_t* dst, cudaStream_t stream);
+
+/* Enqueues a copy of status word 0 of workspace `ws` to `dst` (HOST or device memory, 4 bytes)
+ * on `stream`; see "Device status" above (no counterpart in the paper). */
+MUSE_API int muse_status_copy(const void* ws, int32_t* dst, cudaStream_t stream);
 
 /* Buckets the keys by (cluster, block) and builds the accumulated tilted summaries
  * mu_ijb = log sum exp(sigma qbar_i.k), kappa_ijb, nu_ijb = weighted means of k, v over the
@@ -145,10 +178,15 @@ MUSE_API size_t muse_cluster_noalloc_max_bytes(void);
  *   K, V, assign_k, qbar  in
  *   off_k     out [B,Hkv,Ck*S+1]   bucket offsets
  *   perm_k    out [B,Hkv,N]        bucketed position -> key index
+ *   counts    out [B,Hkv,Ck,S]     keys per bucket (j, b)                 } the untilted
+ *   ksum      out [B,Hkv,Ck,S,D]   fp32 sum of the keys of bucket (j, b)   } per-block statistics
+ *   vsum      out [B,Hkv,Ck,S,D]   fp32 sum of its values                  } (Eq. 3-5 at zero tilt);
+ *                                  pass all three or NULL for all three
  *   summaries out opaque, muse_workspace_bytes out[4] bytes (layout: muse_summaries_layout) */
 MUSE_API int muse_summarize(const muse_params_t* p, const void* K, const void* V,
                    const int32_t* assign_k, const float* qbar,
-                   int32_t* off_k, int32_t* perm_k, void* summaries,
+                   int32_t* off_k, int32_t* perm_k,
+                   int32_t* counts, float* ksum, float* vsum, void* summaries,
                    void* ws, size_t ws_bytes, cudaStream_t stream);
 
 /* Forward: per query, score every key cluster (Eq. 6), retrieve the top-m for exact
@@ -167,6 +205,9 @@ MUSE_API int muse_attn_fwd(const muse_params_t* p, const void* Q, const void* K,
 /* Backward of sum(O * dO) w.r.t. Q, K, V with assign_*, sel and qbar constant; dK, dV of a
  * kv head are summed over the query heads that share it.
  *   O, LSE, sel  in   as returned by muse_attn_fwd (sel must be the selection used there)
+ *   summaries    in   as written by muse_summarize, or NULL: the summaries are then rebuilt from
+ *                     K, V, off_k, perm_k, qbar inside the scratch, which must hold
+ *                     muse_workspace_bytes out[5] bytes instead of out[3]
  *   dQ, dK, dV   out  dtype */
 MUSE_API int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K, const void* V,
                   const void* O, const float* LSE, const void* dO,
@@ -183,6 +224,18 @@ MUSE_API int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K,
  * negative MUSE_ERR_* code.  Not thread-safe with respect to concurrent library calls. */
 MUSE_API int muse_profile(int enable);
 MUSE_API long muse_profile_report(char* buf, size_t cap);
+
+/* Test hooks (no counterpart in the paper; not for production use).
+ * muse_test_force_paths: bit mask; a set bit makes later calls take the library's other kernel
+ *   for one step at shapes where the tensor-core kernel is the default (1 summaries, 2 far field
+ *   forward and backward, 4 key-side summary backward, 8 retrieval forward per (cluster, plane)
+ *   group, 16 retrieval backward as separate dQ and dK/dV kernels, 32 dipole merge, 64 / 128 the
+ *   previous cluster-resident retrieval forward / backward kernels); 0 restores the default.  Process-wide.
+ * muse_test_wait_timeout: clears the status words of `ws` (>= 256 bytes) and launches a one-warp
+ *   kernel whose bounded wait can never be satisfied, with a limit of `limit_clocks` SM clocks:
+ *   word 0 ends up MUSE_STATUS_SELFTEST_TIMEOUT and the context stays usable. */
+MUSE_API int muse_test_force_paths(unsigned mask);
+MUSE_API int muse_test_wait_timeout(void* ws, unsigned limit_clocks, cudaStream_t stream);
 
 /* Human-readable text for a return code (static storage). */
 MUSE_API const char* muse_strerror(int code);

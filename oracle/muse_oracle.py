@@ -472,12 +472,14 @@ def backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=N
     muh, kah, nuh = accumulated_summaries(K, V, a_k, qbar, sigma, S, Ck, causal)
     dQ = np.zeros((N, D)); dK = np.zeros((N, D)); dV = np.zeros((N, Dv))
     dmu = np.zeros_like(muh); dka = np.zeros_like(kah); dnu = np.zeros_like(nuh)
-    fwd = dict(O=np.zeros((N, Dv)), LSE=np.full(N, -np.inf), sel=np.full((N, m), -1, np.int32))
+    fwd = dict(O=np.zeros((N, Dv)), LSE=np.full(N, -np.inf), sel=np.full((N, m), -1, np.int32),
+               sel_gap=np.full(N, np.inf))
     for b, i, r in _segments(a_q, N, S, causal, rows):
         seg = _segment(Q, K, V, a_k, qbar[i], muh[b, i], kah[b, i], nuh[b, i], r, b,
                        sigma=sigma, Bs=Bs, m=m, causal=causal,
                        sel_rows=None if sel is None else sel[r], sel_mode=sel_mode)
         fwd["O"][r], fwd["LSE"][r], fwd["sel"][r] = seg["O"], seg["L"], seg["sel"]
+        fwd["sel_gap"][r] = seg["sel_gap"]
         L = seg["L"][:, None]
         g_out = dO[r]
         delta = (g_out * seg["O"]).sum(1, keepdims=True)

@@ -22,7 +22,12 @@ MUSE_INIT_INDICES, MUSE_INIT_STRIDED, MUSE_INIT_CENTRES = 0, 1, 2
 
 EXPORTS = ("muse_workspace_bytes", "muse_summaries_layout", "muse_cluster", "muse_summarize",
            "muse_attn_fwd", "muse_attn_bwd", "muse_cluster_noalloc", "muse_cluster_noalloc_max_bytes",
-           "muse_profile", "muse_profile_report", "muse_strerror")
+           "muse_cluster_noalloc_status_copy", "muse_status_copy", "muse_test_force_paths",
+           "muse_test_wait_timeout", "muse_profile", "muse_profile_report", "muse_strerror")
+
+# bits of muse_test_force_paths
+FORCE_SUMM_FWD_SIMT, FORCE_FAR_SIMT, FORCE_SUMM_BWD_SIMT, FORCE_RET_FWD_STREAM = 1, 2, 4, 8
+FORCE_RET_BWD_SPLIT, FORCE_DIPOLE_SIMT, FORCE_RET_FWD_OLD, FORCE_RET_BWD_OLD = 16, 32, 64, 128
 
 
 class MuseParams(ctypes.Structure):
@@ -80,12 +85,16 @@ def lib() -> ctypes.CDLL:
         L.muse_workspace_bytes.argtypes = [pp, ctypes.POINTER(sz)]
         L.muse_summaries_layout.argtypes = [pp, ctypes.POINTER(sz)]
         L.muse_cluster.argtypes = [pp, vp, vp, i32p, i32p, i32p, i32p, f32p, f32p, vp, sz, vp]
-        L.muse_summarize.argtypes = [pp, vp, vp, i32p, f32p, i32p, i32p, vp, vp, sz, vp]
+        L.muse_summarize.argtypes = [pp, vp, vp, i32p, f32p, i32p, i32p, i32p, f32p, f32p, vp, vp, sz, vp]
         L.muse_attn_fwd.argtypes = [pp, vp, vp, vp, i32p, f32p, i32p, i32p, vp, i32p, vp, f32p, i32p, vp, sz, vp]
         L.muse_attn_bwd.argtypes = [pp, vp, vp, vp, vp, f32p, vp, i32p, f32p, i32p, i32p, vp, i32p, vp, vp, vp,
                                     vp, sz, vp]
         L.muse_cluster_noalloc.argtypes = [pp, vp, vp, i32p, i32p, i32p, i32p, f32p, f32p, vp]
         L.muse_cluster_noalloc_max_bytes.argtypes = []
+        L.muse_cluster_noalloc_status_copy.argtypes = [vp, vp]
+        L.muse_status_copy.argtypes = [vp, vp, vp]
+        L.muse_test_force_paths.argtypes = [ctypes.c_uint]
+        L.muse_test_wait_timeout.argtypes = [vp, ctypes.c_uint, vp]
         L.muse_profile.argtypes = [ctypes.c_int]
         L.muse_profile_report.argtypes = [ctypes.c_char_p, sz]
         for name in EXPORTS[:-1]:
@@ -117,8 +126,8 @@ def _stream():
 
 
 def muse_workspace_bytes(p: MuseParams):
-    """(cluster, summarize, attn_fwd, attn_bwd, summaries) sizes in bytes."""
-    out = (ctypes.c_size_t * 5)()
+    """(cluster, summarize, attn_fwd, attn_bwd, summaries, attn_bwd without stored summaries) sizes in bytes."""
+    out = (ctypes.c_size_t * 6)()
     _check(lib().muse_workspace_bytes(ctypes.byref(p), out), "muse_workspace_bytes")
     return tuple(int(x) for x in out)
 
@@ -166,10 +175,32 @@ def muse_cluster_noalloc_max_bytes() -> int:
     return int(lib().muse_cluster_noalloc_max_bytes())
 
 
-def muse_summarize(p, K, V, assign_k, qbar, off_k, perm_k, summaries, ws):
+def muse_summarize(p, K, V, assign_k, qbar, off_k, perm_k, summaries, ws, counts=None, ksum=None, vsum=None):
     _check(lib().muse_summarize(ctypes.byref(p), _ptr(K), _ptr(V), _ptr(assign_k), _ptr(qbar), _ptr(off_k),
-                                _ptr(perm_k), _ptr(summaries), _ptr(ws), ws.numel() * ws.element_size(),
-                                _stream()), "muse_summarize")
+                                _ptr(perm_k), _ptr(counts), _ptr(ksum), _ptr(vsum), _ptr(summaries), _ptr(ws),
+                                ws.numel() * ws.element_size(), _stream()), "muse_summarize")
+
+
+def muse_status(ws) -> int:
+    """Status word 0 of a workspace after the stream has drained (0 = every kernel of the last call
+    that used `ws` ran to completion; otherwise a MUSE_STATUS_* code)."""
+    out = torch.zeros(1, dtype=torch.int32, device=ws.device)
+    _check(lib().muse_status_copy(_ptr(ws), _ptr(out), _stream()), "muse_status_copy")
+    return int(out.item())
+
+
+def muse_cluster_noalloc_status() -> int:
+    out = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check(lib().muse_cluster_noalloc_status_copy(_ptr(out), _stream()), "muse_cluster_noalloc_status_copy")
+    return int(out.item())
+
+
+def muse_test_force_paths(mask: int) -> None:
+    _check(lib().muse_test_force_paths(int(mask)), "muse_test_force_paths")
+
+
+def muse_test_wait_timeout(ws, limit_clocks: int) -> None:
+    _check(lib().muse_test_wait_timeout(_ptr(ws), int(limit_clocks), _stream()), "muse_test_wait_timeout")
 
 
 def muse_attn_fwd(p, Q, K, V, assign_q, qbar, off_k, perm_k, summaries, sel_in, O, LSE, sel_out, ws):
@@ -206,6 +237,7 @@ class MuseBuffers:
         self.O = e(B, Hq, N, D, dtype=dt); self.LSE = e(B, Hq, N, dtype=f32)
         self.sel = e(B, Hq, N, max(m, 1), dtype=i32)
         need = max(sizes[:3] + ((sizes[3],) if backward else ()))
+        self.sizes = sizes
         self.ws = e(need, dtype=torch.uint8)
         if backward:
             self.dQ = e(B, Hq, N, D, dtype=dt); self.dK = e(B, Hkv, N, D, dtype=dt); self.dV = e(B, Hkv, N, D, dtype=dt)

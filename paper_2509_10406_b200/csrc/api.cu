@@ -1,11 +1,28 @@
 // C-ABI entry points: argument validation on the host, then the stage launchers.
 #include "common.cuh"
+#include "tc05.cuh"
 
 using namespace muse;
 
 namespace {
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+unsigned g_forced_paths = 0;
+
+// The status words are cleared once per public call (every kernel of the call reports into them).
+int clear_status(void* ws, cudaStream_t st) {
+  return cudaMemsetAsync(ws, 0, kStatusWords * sizeof(int32_t), st) == cudaSuccess ? MUSE_OK : MUSE_ERR_CUDA;
+}
+
+// A deliberately unreachable wait: nothing ever arrives at the barrier, so the bounded wait runs out
+// after `limit_clocks` and the kernel reports through the status word like any production kernel.
+__global__ void k_selftest_wait(int* status, unsigned limit_clocks) {
+  __shared__ uint64_t bar;
+  if (threadIdx.x == 0) { tc::mbar_init(&bar, 1); tc::mbar_init_fence(); }
+  __syncthreads();
+  if (threadIdx.x == 0 && !tc::mbar_wait(&bar, 0, limit_clocks)) report_status(status, MUSE_STATUS_SELFTEST_TIMEOUT);
+}
 
 // Validates the parameter block and resolves defaults.  Returns MUSE_OK or an error code.
 int resolve(const muse_params_t* p, Dims* d) {
@@ -45,7 +62,25 @@ int resolve(const muse_params_t* p, Dims* d) {
 
 }  // namespace
 
+namespace muse { bool path_forced(unsigned bit) { return (g_forced_paths & bit) != 0; } }
+
 extern "C" {
+
+int muse_test_force_paths(unsigned mask) { g_forced_paths = mask; return MUSE_OK; }
+
+int muse_status_copy(const void* ws, int32_t* dst, cudaStream_t stream) {
+  if (ws == nullptr || dst == nullptr) return MUSE_ERR_INVALID_ARG;
+  MUSE_CUDA_OK(cudaMemcpyAsync(dst, ws, sizeof(int32_t), cudaMemcpyDefault, stream));
+  return MUSE_OK;
+}
+
+int muse_test_wait_timeout(void* ws, unsigned limit_clocks, cudaStream_t stream) {
+  if (ws == nullptr) return MUSE_ERR_INVALID_ARG;
+  if (clear_status(ws, stream) != MUSE_OK) return MUSE_ERR_CUDA;
+  k_selftest_wait<<<1, 32, 0, stream>>>((int*)ws, limit_clocks);
+  MUSE_LAUNCH_OK();
+  return MUSE_OK;
+}
 
 const char* muse_strerror(int code) {
   switch (code) {
@@ -58,7 +93,7 @@ const char* muse_strerror(int code) {
   }
 }
 
-int muse_workspace_bytes(const muse_params_t* p, size_t out[5]) {
+int muse_workspace_bytes(const muse_params_t* p, size_t out[6]) {
   Dims d;
   int rc = resolve(p, &d);
   if (rc != MUSE_OK) return rc;
@@ -70,6 +105,8 @@ int muse_workspace_bytes(const muse_params_t* p, size_t out[5]) {
   out[3] = attn_bwd_ws_bytes(d, p->dtype);
   out[4] = summ_layout(d, p->dtype).total;
   for (int k = 0; k < 4; ++k) if (out[k] < 256) out[k] = 256;
+  // backward without stored summaries: its scratch, then a summaries buffer, then the summaries stage's scratch
+  out[5] = out[3] + out[4] + out[1];
   return MUSE_OK;
 }
 
@@ -91,9 +128,10 @@ int muse_cluster(const muse_params_t* p, const void* Q, const void* K, const int
   if (rc != MUSE_OK) return rc;
   if (ws == nullptr || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;
   if (Q == nullptr && K == nullptr) return MUSE_ERR_INVALID_ARG;
-  size_t need[5];
+  size_t need[6];
   muse_workspace_bytes(p, need);
   if (ws_bytes < need[0]) return MUSE_ERR_WORKSPACE;
+  if (clear_status(ws, stream) != MUSE_OK) return MUSE_ERR_CUDA;
   if (Q != nullptr) {
     if (assign_q == nullptr || qbar == nullptr || !aligned16(Q) || !aligned16(qbar)) return MUSE_ERR_INVALID_ARG;
     if (p->init_mode == MUSE_INIT_INDICES && init_q == nullptr) return MUSE_ERR_INVALID_ARG;
@@ -111,17 +149,21 @@ int muse_cluster(const muse_params_t* p, const void* Q, const void* K, const int
 }
 
 int muse_summarize(const muse_params_t* p, const void* K, const void* V, const int32_t* assign_k,
-                   const float* qbar, int32_t* off_k, int32_t* perm_k, void* summaries, void* ws,
-                   size_t ws_bytes, cudaStream_t stream) {
+                   const float* qbar, int32_t* off_k, int32_t* perm_k, int32_t* counts, float* ksum, float* vsum,
+                   void* summaries, void* ws, size_t ws_bytes, cudaStream_t stream) {
   Dims d;
   int rc = resolve(p, &d);
   if (rc != MUSE_OK) return rc;
   if (!K || !V || !assign_k || !qbar || !off_k || !perm_k || !summaries || !ws) return MUSE_ERR_INVALID_ARG;
   if (!aligned16(K) || !aligned16(V) || !aligned16(qbar) || !aligned16(summaries) || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;
-  size_t need[5];
+  const int nstat = (counts != nullptr) + (ksum != nullptr) + (vsum != nullptr);
+  if (nstat != 0 && nstat != 3) return MUSE_ERR_INVALID_ARG;            // the three untilted outputs come together
+  if (nstat == 3 && (!aligned16(ksum) || !aligned16(vsum))) return MUSE_ERR_INVALID_ARG;
+  size_t need[6];
   muse_workspace_bytes(p, need);
   if (ws_bytes < need[1]) return MUSE_ERR_WORKSPACE;
-  rc = summarize(d, p->dtype, K, V, assign_k, qbar, off_k, perm_k, summaries, ws, stream);
+  if (clear_status(ws, stream) != MUSE_OK) return MUSE_ERR_CUDA;
+  rc = summarize(d, p->dtype, K, V, assign_k, qbar, off_k, perm_k, counts, ksum, vsum, summaries, ws, nullptr, stream);
   prof_mark(nullptr, stream);
   return rc;
 }
@@ -135,9 +177,10 @@ int muse_attn_fwd(const muse_params_t* p, const void* Q, const void* K, const vo
   if (rc != MUSE_OK) return rc;
   if (!Q || !K || !V || !assign_q || !qbar || !off_k || !perm_k || !summaries || !O || !LSE || !ws) return MUSE_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(qbar) || !aligned16(summaries) || !aligned16(O) || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;
-  size_t need[5];
+  size_t need[6];
   muse_workspace_bytes(p, need);
   if (ws_bytes < need[2]) return MUSE_ERR_WORKSPACE;
+  if (clear_status(ws, stream) != MUSE_OK) return MUSE_ERR_CUDA;
   rc = attn_fwd(d, p->dtype, Q, K, V, assign_q, qbar, off_k, perm_k, summaries, sel_in, O, LSE, sel_out, ws, stream);
   prof_mark(nullptr, stream);
   return rc;
@@ -150,14 +193,24 @@ int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K, const vo
   Dims d;
   int rc = resolve(p, &d);
   if (rc != MUSE_OK) return rc;
-  if (!Q || !K || !V || !O || !LSE || !dO || !assign_q || !qbar || !off_k || !perm_k || !summaries || !dQ || !dK || !dV || !ws) return MUSE_ERR_INVALID_ARG;
+  if (!Q || !K || !V || !O || !LSE || !dO || !assign_q || !qbar || !off_k || !perm_k || !dQ || !dK || !dV || !ws) return MUSE_ERR_INVALID_ARG;
   if (d.dipole) return MUSE_ERR_UNSUPPORTED;       // no backward through the dipole correction
   if (d.m > 0 && d.SB > 0 && sel == nullptr) return MUSE_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(qbar) ||
       !aligned16(summaries) || !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;
-  size_t need[5];
+  size_t need[6];
   muse_workspace_bytes(p, need);
-  if (ws_bytes < need[3]) return MUSE_ERR_WORKSPACE;
+  if (ws_bytes < (summaries ? need[3] : need[5])) return MUSE_ERR_WORKSPACE;
+  if (clear_status(ws, stream) != MUSE_OK) return MUSE_ERR_CUDA;
+  if (summaries == nullptr) {
+    // Rebuild the summaries from the bucketed keys in the tail of the workspace (the keys keep the
+    // bucketing that off_k / perm_k describe, so no sort is needed).
+    char* tail = (char*)ws + need[3];
+    rc = summarize(d, p->dtype, K, V, nullptr, qbar, const_cast<int32_t*>(off_k), const_cast<int32_t*>(perm_k), nullptr, nullptr,
+                   nullptr, tail, tail + need[4], (int32_t*)ws, stream);
+    if (rc != MUSE_OK) return rc;
+    summaries = tail;
+  }
   rc = attn_bwd(d, p->dtype, Q, K, V, O, LSE, dO, assign_q, qbar, off_k, perm_k, summaries, sel, dQ, dK, dV, ws, stream);
   prof_mark(nullptr, stream);
   return rc;

@@ -130,10 +130,11 @@ k_assign_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
       const float ob = best_s[row];
       const int oi = idx_s[row];
       if (ob < best || (ob == best && oi < bidx)) bidx = oi;
-      if (row0 + row < N) assign[(size_t)prob * N + row0 + row] = bidx;
+      // a row of NaN or infinities never compares below the running minimum: it goes to cluster 0
+      if (row0 + row < N) assign[(size_t)prob * N + row0 + row] = (unsigned)bidx < (unsigned)C ? bidx : 0;
     }
   }
-  if (!ok) atomicExch(status, 6);
+  if (!ok) report_status(status, 6);
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tbase, 2 * kAtCols);

@@ -5,7 +5,6 @@
 // (Appendix "Aggregation Weight Gradient Flow").
 #include "common.cuh"
 #include "flash_core.cuh"
-#include <cstdlib>
 
 namespace muse {
 
@@ -597,7 +596,8 @@ __global__ void k_final_dq(Dims dm, const float* __restrict__ dQacc, const PT* _
   for (int k = 0; k < D / 32; ++k) acc[k] = dQacc[row * D + lane + 32 * k];
   if (use_ret && query_plane_b(dm, t) >= 0) {
     for (int s = 0; s < dm.m; ++s) {
-      if (sel[row * dm.m + s] < 0) continue;
+      const int c = sel[row * dm.m + s];
+      if (c < 0 || c >= dm.Ck) continue;                   // "none", or an entry outside [0, Ck), which counts as none
 #pragma unroll
       for (int k = 0; k < D / 32; ++k) acc[k] += to_f(dq_part[(row * dm.m + s) * D + lane + 32 * k]);
     }
@@ -701,7 +701,6 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
   MUSE_CUDA_OK(cudaMemsetAsync(w.dV_perm, 0, nd, st));
   const size_t sm4 = 4 * tile_bytes<T, D>() + ptile_bytes();
   constexpr bool kTensor = sizeof(T) == 2;      // bf16 mode runs the exact-attention parts on tcgen05
-  MUSE_CUDA_OK(cudaMemsetAsync(w.status, 0, 64 * sizeof(int32_t), st));
   if (d.causal && kTensor) {
     int rc = local_bwd_tc(d, Q, K, V, dO, LSE, w.delta, w.dQacc, w.dK_orig, w.dV_orig, w.status, st);
     if (rc != MUSE_OK) return rc;
@@ -739,9 +738,9 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
       }
       use_ret = 1;
     }
-    const bool far_tc = far_bwd_tc_supported(d, dtype) && getenv("MUSE_FAR_SIMT") == nullptr;
+    const bool far_tc = far_bwd_tc_supported(d, dtype) && !path_forced(kForceFarSimt);
     const size_t fsm = (size_t)(4 * kTile * (D + 4) + kTile * kLDP) * sizeof(float) + (size_t)kTile * cdiv(d.Ck, 32) * sizeof(uint32_t);
-    const bool summ_tc = far_tc && summ_bwd_tc_supported(d, dtype) && getenv("MUSE_SUMM_SIMT") == nullptr;
+    const bool summ_tc = far_tc && summ_bwd_tc_supported(d, dtype) && !path_forced(kForceSummBwdSimt);
     if (far_tc) {
       rc = far_bwd_tc(d, sp, Q, dO, qbar, LSE, w.delta, w.off_q, w.perm_q, sel, w.dQacc, w.dkappa, w.dnu, w.dS, summ_tc ? 1 : 0, w.status, st);
       if (rc != MUSE_OK) return rc;

@@ -12,7 +12,6 @@
 #include "common.cuh"
 #include "tc05.cuh"
 
-#include <cstdlib>
 
 namespace muse {
 
@@ -87,7 +86,7 @@ __device__ __forceinline__ void bwd_teardown(BwdCtx& c, uint32_t cols, int tid, 
   tc::fence_before_sync();
   __syncthreads();
   if ((tid >> 5) == 0) tc::tmem_dealloc(c.tbase, cols);
-  if (!c.ok && tid == 0) atomicExch(status, 2);
+  if (!c.ok && tid == 0) report_status(status, 2);
 }
 
 __device__ __forceinline__ void store_row64(unsigned char* tile, int row, const float (&x)[kBN]) {
@@ -631,7 +630,7 @@ k_local_bwd_dkdv_tc(Dims dm, const __grid_constant__ CUtensorMap tm_q, const __g
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tbase, SM::cols);
-  if (!ok && tid == 0) atomicExch(status, 2);
+  if (!ok && tid == 0) report_status(status, 2);
 }
 
 // One CTA per (key cluster j, plane, split, head): 128-key tiles of the run the plane sees, fed with
@@ -805,7 +804,7 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   const int nsub = min(kFusedSplit, max(1, ntiles_all / kFusedTilesPerCta));
   if (ntiles_all == 0 || sub >= nsub) return;
   if (tc::smem_u32(sm_raw) & 1023u) {                      // the tiles fill the whole dynamic allocation: no room to realign
-    if (tid == 0) atomicExch(status, 2);
+    if (tid == 0) report_status(status, 2);
     return;
   }
   if (tid == 0) { err_s = 0; tc::mbar_init(&bar_rows[0], kFusedGather); tc::mbar_init(&bar_rows[1], kFusedGather); }
@@ -1154,7 +1153,7 @@ int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, con
                const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, void* dq_part,
                float* dK_perm, float* dV_perm, int* status, cudaStream_t st) {
   const int pq = d.B * d.Hq;
-  if (d.D == 128 && getenv("MUSE_RET_BWD_SPLIT") == nullptr) {
+  if (d.D == 128 && !path_forced(kForceRetBwdSplit)) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_bwd_fused_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, FusedSmem::total));
     prof_mark("k_ret_bwd_fused_tc", st);
     k_ret_bwd_fused_tc<<<dim3(d.Ck, kFusedSplit, pq), kFusedThreads, FusedSmem::total, st>>>(d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp, (const bf16*)Vp,

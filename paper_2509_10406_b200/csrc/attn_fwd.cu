@@ -4,7 +4,6 @@
 // and the log-sum-exp merge ("Output merging").
 #include "common.cuh"
 #include "flash_core.cuh"
-#include <cstdlib>
 
 namespace muse {
 
@@ -22,8 +21,8 @@ int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, con
 __device__ __forceinline__ int query_plane(const Dims& d, int t) { return d.causal ? t / d.Bs - 1 : 0; }
 
 // ---------------------------------------------------------------------------------------------
-// Inverse index for retrieval (Section "Exact retrieval": "an inverse index mapping each
-// (cluster, block) to the queries that retrieve it").  Group key = plane * Ck + cluster.
+// Inverse index for retrieval (Section "Exact Retrieval and Local Attention"): for every
+// (plane, key cluster) the list of (query, slot) pairs that retrieve it.  Group key = plane * Ck + cluster.
 // ---------------------------------------------------------------------------------------------
 // Thread e handles (slot = e / N, query = e % N): the lanes of a warp are consecutive queries,
 // which often retrieve the same cluster in the same slot, so equal keys are combined with a warp
@@ -36,7 +35,7 @@ __global__ void k_ret_count(Dims d, const int32_t* __restrict__ sel, int32_t* __
     const int t = (int)(e % d.N), k = (int)(e / d.N);
     const int c = sel[((size_t)pq * d.N + t) * d.m + k];
     const int pl = query_plane(d, t);
-    if (c >= 0 && pl >= 0) key = pl * d.Ck + c;
+    if (c >= 0 && c < d.Ck && pl >= 0) key = pl * d.Ck + c;      // entries outside [0, Ck) count as "none"
   }
   const unsigned peers = __match_any_sync(0xffffffffu, key);
   const int lane = threadIdx.x & 31;
@@ -52,7 +51,7 @@ __global__ void k_ret_fill(Dims d, const int32_t* __restrict__ sel, int32_t* __r
     const int t = (int)(e % d.N), k = (int)(e / d.N);
     const int c = sel[((size_t)pq * d.N + t) * d.m + k];
     const int pl = query_plane(d, t);
-    if (c >= 0 && pl >= 0) { key = pl * d.Ck + c; pid = t * d.m + k; }
+    if (c >= 0 && c < d.Ck && pl >= 0) { key = pl * d.Ck + c; pid = t * d.m + k; }
   }
   const unsigned peers = __match_any_sync(0xffffffffu, key);
   const int lane = threadIdx.x & 31, leader = __ffs(peers) - 1;
@@ -203,7 +202,7 @@ k_far_fwd(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, cons
       int32_t* so = sel_out + ((size_t)pq * dm.N + t) * m;
       if (sel_in != nullptr) {
         const int32_t* si = sel_in + ((size_t)pq * dm.N + t) * m;
-        for (int k = lane; k < m; k += 32) { int c = si[k]; so[k] = c; if (c >= 0 && c < Ck) s[c] = -INFINITY; }
+        for (int k = lane; k < m; k += 32) { int c = si[k]; c = (c >= 0 && c < Ck) ? c : -1; so[k] = c; if (c >= 0) s[c] = -INFINITY; }
       } else if (dm.sel_mode == MUSE_SEL_PER_QCLUSTER) {
         for (int k = lane; k < m; k += 32) { int c = selq[k]; so[k] = c; if (c >= 0) s[c] = -INFINITY; }
       } else {
@@ -550,7 +549,6 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
   int32_t* sel = sel_out ? sel_out : w.sel_tmp;
   const size_t fl_smem = 3 * tile_bytes<T, D>() + ptile_bytes();
   constexpr bool kTensor = sizeof(T) == 2;      // bf16 mode runs the exact-attention parts on tcgen05
-  MUSE_CUDA_OK(cudaMemsetAsync(w.status, 0, 64 * sizeof(int32_t), st));
   // local attention
   if (d.causal && kTensor) {
     int rc = local_fwd_tc(d, Q, K, V, w.o_loc, w.lse_loc, w.status, st);
@@ -567,7 +565,7 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
   if (d.SB > 0) {
     int rc = bucket_sort(0, assign_q, pq, d.N, d.Cq, d.S, d.Bs, 0, w.off_q, w.perm_q, w.sort_scratch, st);
     if (rc != MUSE_OK) return rc;
-    if (far_fwd_tc_supported(d, dtype) && getenv("MUSE_FAR_SIMT") == nullptr) {
+    if (far_fwd_tc_supported(d, dtype) && !path_forced(kForceFarSimt)) {
       rc = far_fwd_tc(d, summ_ptrs(L, base), Q, w.off_q, w.perm_q, sel_in, sel, w.o_far, w.lse_far, w.status, st);
       if (rc != MUSE_OK) return rc;
     } else {

@@ -9,7 +9,6 @@
 #include "common.cuh"
 #include "tc05.cuh"
 
-#include <cstdlib>
 
 namespace muse {
 
@@ -163,7 +162,7 @@ __device__ __forceinline__ void tc_teardown(TcCtx& c, int tid, int* status) {
   tc::fence_before_sync();
   __syncthreads();
   if ((tid >> 5) == 0) tc::tmem_dealloc(c.tbase, D == 128 ? 256 : 128);
-  if (!c.ok && tid == 0) atomicExch(status, 1);
+  if (!c.ok && tid == 0) report_status(status, 1);
 }
 
 // ---- local (block-diagonal) attention ------------------------------------------------------------
@@ -350,7 +349,7 @@ k_local_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_k, const __grid_c
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tbase, 256);
-  if (!ok && tid == 0) atomicExch(status, 1);
+  if (!ok && tid == 0) report_status(status, 1);
 }
 
 // ---- exact retrieval ---------------------------------------------------------------------------------
@@ -796,7 +795,7 @@ k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tbase, SM::cols);
-  if (!ok_ && tid == 0) atomicExch(status, 1);
+  if (!ok_ && tid == 0) report_status(status, 1);
 }
 
 int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
@@ -825,7 +824,7 @@ int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, con
                const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st) {
   dim3 grid(d.Ck, d.SB * kRetFwdSplit, d.B * d.Hq);
   const int min_keys = 0;
-  if (d.D == 128 && getenv("MUSE_RET_FWD_STREAM") == nullptr) {
+  if (d.D == 128 && !path_forced(kForceRetFwdStream)) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_cluster_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, RcSmem::total));
     prof_mark("k_ret_fwd_cluster_tc", st);
     k_ret_fwd_cluster_tc<<<dim3(d.Ck, kRcSplit, d.B * d.Hq), kRcThreads, RcSmem::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k,

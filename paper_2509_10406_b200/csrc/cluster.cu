@@ -16,6 +16,7 @@ constexpr int kSortThreads = 256;
 
 __device__ __forceinline__ int sort_key(int t, int a, int C, int S, int Bs, int kind) {
   int b = t / Bs;
+  a = min(max(a, 0), C - 1);             // a caller-provided assignment outside [0, C) is pinned, never used as an index
   return kind == 0 ? b * C + a : a * S + b;
 }
 
@@ -314,7 +315,8 @@ k_assign(const T* __restrict__ X, int N, int C, const float* __restrict__ centre
       if (ob < b || (ob == b && oi < i)) { b = ob; i = oi; }
     }
     int row = row0 + ty * 8 + r;
-    if (tx == 0 && row < N) assign[(size_t)prob * N + row] = i;
+    // a row of NaN or infinities never compares below the running minimum: it goes to cluster 0
+    if (tx == 0 && row < N) assign[(size_t)prob * N + row] = (unsigned)i < (unsigned)C ? i : 0;
   }
 }
 
@@ -373,7 +375,7 @@ static int lloyd_t(const Dims& d, const T* X, int problems, int C, int kind, con
                    int init_mode, uint64_t seed, int T_iters, int32_t* assign, float* centres, void* ws,
                    cudaStream_t st) {
   Arena ar(ws);
-  int32_t* status = ar.take<int32_t>(64);      // ws[0]: non-zero if a bounded device-side wait gave up
+  int32_t* status = ar.take<int32_t>(kStatusWords);     // cleared by the entry point, shared by both sides
   float* cnorm = ar.take<float>((size_t)problems * C);
   int32_t* off = ar.take<int32_t>((size_t)problems * (C * d.S + 1));
   int32_t* perm = ar.take<int32_t>((size_t)problems * d.N);
@@ -381,7 +383,6 @@ static int lloyd_t(const Dims& d, const T* X, int problems, int C, int kind, con
   __nv_bfloat16* chi = ar.take<__nv_bfloat16>((size_t)problems * C * D);
   __nv_bfloat16* clo = ar.take<__nv_bfloat16>((size_t)problems * C * D);
   constexpr bool kTensor = sizeof(T) == 2;     // bf16 inputs: distances on the tensor cores
-  MUSE_CUDA_OK(cudaMemsetAsync(status, 0, 64 * sizeof(int32_t), st));
   if (init_mode != MUSE_INIT_CENTRES) {
     prof_mark("k_init_centres", st);
     k_init_centres<T><<<dim3(C, problems), 32, 0, st>>>(X, d.N, D, C, init_idx, init_mode, seed, kind, centres);

@@ -10,20 +10,19 @@ namespace {
 constexpr size_t kStaticScratchBytes = size_t(32) << 20;
 static __device__ __align__(256) unsigned char g_cluster_scratch[kStaticScratchBytes];
 
-// In host code `g_cluster_scratch` is only a stand-in for the symbol, not a device address:
-// the address is looked up once per device, with that device current.
-constexpr int kMaxDevices = 64;
-void* g_scratch_addr[kMaxDevices] = {nullptr};
-
+// In host code `g_cluster_scratch` is only a stand-in for the symbol, not a device address.
+// The address is looked up on every call, with the caller's device current: once the module is
+// loaded on that device this is a cheap host-side lookup, and nothing is cached that a device
+// reset or a new primary context could leave stale.  The very first lookup on a device loads the
+// library's device image there, which is when the 32 MiB are actually reserved (and the one
+// point where this entry can fail for lack of memory).
 int scratch_address(void** out) {
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MUSE_ERR_CUDA;
-  if (g_scratch_addr[dev] == nullptr) {
-    void* p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_cluster_scratch) != cudaSuccess || p == nullptr) return MUSE_ERR_CUDA;
-    g_scratch_addr[dev] = p;
+  void* p = nullptr;
+  if (cudaGetSymbolAddress(&p, g_cluster_scratch) != cudaSuccess || p == nullptr) {
+    cudaGetLastError();                                    // leave no sticky error for the next launch check
+    return MUSE_ERR_CUDA;
   }
-  *out = g_scratch_addr[dev];
+  *out = p;
   return MUSE_OK;
 }
 
@@ -36,7 +35,7 @@ size_t muse_cluster_noalloc_max_bytes(void) { return kStaticScratchBytes; }
 int muse_cluster_noalloc(const muse_params_t* p, const void* Q, const void* K, const int32_t* init_q,
                          const int32_t* init_k, int32_t* assign_q, int32_t* assign_k, float* qbar, float* kcent,
                          cudaStream_t stream) {
-  size_t need[5];
+  size_t need[6];
   int rc = muse_workspace_bytes(p, need);
   if (rc != MUSE_OK) return rc;
   if (need[0] > kStaticScratchBytes) return MUSE_ERR_WORKSPACE;    // problem too large for the built-in scratch
@@ -47,6 +46,18 @@ int muse_cluster_noalloc(const muse_params_t* p, const void* Q, const void* K, c
   // what the stage already clears itself (its status words and its shared-memory histograms;
   // the sort counters are fully rewritten before they are read).
   return muse_cluster(p, Q, K, init_q, init_k, assign_q, assign_k, qbar, kcent, ws, kStaticScratchBytes, stream);
+}
+
+
+// The status word of the last muse_cluster_noalloc call lives inside the built-in array, where the
+// caller cannot point: this enqueues its 4-byte copy to `dst` (host or device memory) on `stream`.
+int muse_cluster_noalloc_status_copy(int32_t* dst, cudaStream_t stream) {
+  if (dst == nullptr) return MUSE_ERR_INVALID_ARG;
+  void* ws = nullptr;
+  int rc = scratch_address(&ws);
+  if (rc != MUSE_OK) return rc;
+  MUSE_CUDA_OK(cudaMemcpyAsync(dst, ws, sizeof(int32_t), cudaMemcpyDefault, stream));
+  return MUSE_OK;
 }
 
 }  // extern "C"

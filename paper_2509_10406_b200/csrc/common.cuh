@@ -100,6 +100,20 @@ __device__ __forceinline__ float warp_max(float v) {
 // per-kernel timing hook (no-op unless muse_profile(1) was called); name = nullptr ends a call
 void prof_mark(const char* name, cudaStream_t st);
 
+// Status words: the first kStatusWords int32 of every stage's workspace.  Word 0 holds the first
+// MUSE_STATUS_* code a kernel reported (0 = none); the entry points clear the words once per call.
+// Words from 8 up carry diagnostics of instrumented builds only.
+constexpr int kStatusWords = 64;
+__device__ __forceinline__ void report_status(int* status, int code) { atomicCAS(status, 0, code); }
+
+// Test hook: bit set = take the library's other kernel for that step at shapes where the default is
+// the tensor-core kernel (muse_test_force_paths; never set in production).
+enum ForcePath : unsigned {
+  kForceSummFwdSimt = 1u, kForceFarSimt = 2u, kForceSummBwdSimt = 4u, kForceRetFwdStream = 8u,
+  kForceRetBwdSplit = 16u, kForceDipoleSimt = 32u, kForceRetFwdOld = 64u, kForceRetBwdOld = 128u
+};
+bool path_forced(unsigned bit);
+
 // ---- stage launchers (each enqueues on `st`, returns MUSE_OK or MUSE_ERR_CUDA) ---------------
 // clustering side: kind 0 = queries (key = block*C + cluster), kind 1 = keys (key = cluster*S + block)
 size_t sort_ws_elems(int N, int nkeys);   // int32 scratch elements per problem for bucket_sort
@@ -111,9 +125,11 @@ int lloyd(const Dims& d, int dtype, const void* X, int problems, int C, int kind
           int32_t* assign, float* centres, void* ws, cudaStream_t st);
 size_t lloyd_ws_bytes(const Dims& d, int problems, int C, int kind);
 
+// assign_k == nullptr: the keys are already bucketed (off_k, perm_k are inputs) and `status` names the
+// caller's status words; counts / ksum / vsum (untilted per-bucket statistics) may be nullptr
 int summarize(const Dims& d, int dtype, const void* K, const void* V, const int32_t* assign_k,
-              const float* qbar, int32_t* off_k, int32_t* perm_k, void* summaries, void* ws,
-              cudaStream_t st);
+              const float* qbar, int32_t* off_k, int32_t* perm_k, int32_t* counts, float* ksum, float* vsum,
+              void* summaries, void* ws, int32_t* status, cudaStream_t st);
 size_t summarize_ws_bytes(const Dims& d, int dtype);
 
 // sigma * qbar as two bf16 planes (hi + lo keeps ~16 mantissa bits), [B*Hq*Cq][D] each: the tensor-core

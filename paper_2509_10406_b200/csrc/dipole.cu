@@ -8,7 +8,6 @@
 //   4. o_far_t += Cbar_ib * sigma (q_t - qbar_i)   (value shift only; the mass is unchanged)
 #include "common.cuh"
 
-#include <cstdlib>
 
 namespace muse {
 
@@ -217,7 +216,7 @@ static int dipole_build_t(const Dims& d, int dtype, const T* Kp, const T* Vp, co
   prof_mark("k_dipole_weights", st);
   k_dipole_weights<ST><<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(mu, rows, d.Ck, P);
   MUSE_LAUNCH_OK();
-  if (dipole_merge_tc_supported(d, dtype) && getenv("MUSE_DIPOLE_SIMT") == nullptr)
+  if (dipole_merge_tc_supported(d, dtype) && !path_forced(kForceDipoleSimt))
     return dipole_merge_tc(d, P, cov, cbar, status, st);
   prof_mark("k_dipole_merge", st);
   k_dipole_merge<ST><<<dim3(D * D / 256, cdiv(d.Cq, kMrgI), d.B * d.Hq * d.SB), 256, 0, st>>>(d, P, cov, cbar);

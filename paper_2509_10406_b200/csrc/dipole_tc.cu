@@ -111,7 +111,7 @@ k_dipole_merge_tc(Dims dm, const __grid_constant__ CUtensorMap tm_p, const __gri
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tbase, kDmCols);
-  if (!ok && tid == 0) atomicExch(status, 7);
+  if (!ok && tid == 0) report_status(status, 7);
 }
 
 bool dipole_merge_tc_supported(const Dims& d, int dtype) {

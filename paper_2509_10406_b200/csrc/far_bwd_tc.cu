@@ -12,7 +12,6 @@
 #include "common.cuh"
 #include "tc05.cuh"
 
-#include <cstdlib>
 
 namespace muse {
 
@@ -404,7 +403,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   __syncthreads();
   if (tid == ISSUER) tc::tma_store_wait_read();             // the staging tiles must outlive the stores' reads only
   if (warp == 0) tc::tmem_dealloc(tbase, 512);
-  if (!ok && tid == 0) atomicExch(status, 4);
+  if (!ok && tid == 0) report_status(status, 4);
 #ifdef MUSE_PHASE_CLOCKS
   if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 3 && blockIdx.z == 0) {
     status[56] = (int)(t_loop_ - t_in_); status[57] = (int)(t_end_ - t_loop_); status[58] = (int)(clock64() - t_end_);

@@ -416,7 +416,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
         int32_t* so = sel_out + ((size_t)pq * dm.N + t) * m;
         if (sel_in != nullptr) {
           const int32_t* si = sel_in + ((size_t)pq * dm.N + t) * m;
-          for (int k = lane; k < m; k += 32) { int c = si[k]; so[k] = c; if (c >= 0 && c < Ck) s[c] = -INFINITY; }
+          for (int k = lane; k < m; k += 32) { int c = si[k]; c = (c >= 0 && c < Ck) ? c : -1; so[k] = c; if (c >= 0) s[c] = -INFINITY; }
         } else if (dm.sel_mode == MUSE_SEL_PER_QCLUSTER) {
           for (int k = lane; k < m; k += 32) { int c = selq[k]; so[k] = c; if (c >= 0) s[c] = -INFINITY; }
         } else if (m > 0) {
@@ -540,7 +540,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tbase, kFarTcCols);
-  if (!ok && tid == 0) atomicExch(status, 3);
+  if (!ok && tid == 0) report_status(status, 3);
 }
 
 bool far_fwd_tc_supported(const Dims& d, int dtype) {

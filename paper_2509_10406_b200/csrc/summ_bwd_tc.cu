@@ -266,7 +266,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
 #ifdef MUSE_PHASE_CLOCKS
   if (tid == 0 && blockIdx.x == 5 && blockIdx.y == 0) for (int k = 0; k < 8; ++k) status[56 + k] = (int)pc[k];
 #endif
-  if (!ok && tid == 0) atomicExch(status, 5);
+  if (!ok && tid == 0) report_status(status, 5);
 }
 
 bool summ_bwd_tc_supported(const Dims& d, int dtype) {

@@ -3,7 +3,6 @@
 // and Causal Accumulation", Eq. 3-5; Algorithm 1 "Causal accumulation along spatial axis").
 #include "common.cuh"
 
-#include <cstdlib>
 
 namespace muse {
 
@@ -40,6 +39,34 @@ __global__ void k_gather_rows(const T* __restrict__ in, const int32_t* __restric
   const uint4* src = reinterpret_cast<const uint4*>(in + ((size_t)prob * N + perm[(size_t)prob * N + p]) * D);
   uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)prob * N + p) * D);
   dst[v] = src[v];
+}
+
+// Untilted per-bucket statistics (Section "Summary Computation": the zero-tilt case of Eq. 3-5):
+// counts n_jb and the plain sums of the keys and of the values of bucket (j, b).  One warp per
+// bucket walks its rows of the bucketed copies in order (fixed summation order).
+template <class T, int D>
+__global__ void k_bucket_sums(const T* __restrict__ Kp, const T* __restrict__ Vp, const int32_t* __restrict__ off_k, int N,
+                              int nbuckets, int32_t* __restrict__ counts, float* __restrict__ ksum, float* __restrict__ vsum) {
+  const int prob = blockIdx.y, lane = threadIdx.x & 31;
+  const int bk = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (bk >= nbuckets) return;
+  const int32_t* o = off_k + (size_t)prob * (nbuckets + 1) + bk;
+  const int p0 = o[0], p1 = o[1];
+  constexpr int EPL = D / 32;
+  float ak[EPL], av[EPL];
+#pragma unroll
+  for (int k = 0; k < EPL; ++k) ak[k] = av[k] = 0.f;
+  for (int p = p0; p < p1; ++p) {
+    float x[EPL], y[EPL];
+    ldv<EPL>(Kp + ((size_t)prob * N + p) * D + lane * EPL, x);
+    ldv<EPL>(Vp + ((size_t)prob * N + p) * D + lane * EPL, y);
+#pragma unroll
+    for (int k = 0; k < EPL; ++k) { ak[k] += x[k]; av[k] += y[k]; }
+  }
+  const size_t e = (size_t)prob * nbuckets + bk;
+  stv<EPL>(ksum + e * D + lane * EPL, ak);
+  stv<EPL>(vsum + e * D + lane * EPL, av);
+  if (lane == 0) counts[e] = p1 - p0;
 }
 
 // One CTA = (key cluster j, tile of 64 query clusters, query head).  It walks the cluster's
@@ -172,12 +199,19 @@ template <class T, int D>
 static int summarize_planes(const Dims& d, int dtype, const T* Kp, const T* Vp, const int32_t* off_k, const float* qbar,
                             const SummLayout& L, char* base, void* qsplit, int32_t* status, cudaStream_t st);
 
+// assign_k == nullptr: off_k and perm_k are inputs (the keys are already bucketed: the backward pass
+// rebuilding the summaries it was not given); `status` then points at the caller's status words.
 template <class T, int D>
 static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const int32_t* assign_k,
-                       const float* qbar, int32_t* off_k, int32_t* perm_k, void* summaries, void* ws,
-                       cudaStream_t st) {
+                       const float* qbar, int32_t* off_k, int32_t* perm_k, int32_t* counts, float* ksum, float* vsum,
+                       void* summaries, void* ws, int32_t* status_in, cudaStream_t st) {
   const int pk = d.B * d.Hkv;
-  int rc = bucket_sort(0, assign_k, pk, d.N, d.Ck, d.S, d.Bs, 1, off_k, perm_k, (int32_t*)ws, st);
+  Arena ar(ws);
+  int32_t* status = ar.take<int32_t>(kStatusWords);      // cleared by the entry point
+  if (status_in != nullptr) status = status_in;
+  int32_t* sort_scratch = ar.take<int32_t>(sort_ws_elems(d.N, d.Ck * d.S) * (size_t)pk);
+  int rc = MUSE_OK;
+  if (assign_k != nullptr) rc = bucket_sort(0, assign_k, pk, d.N, d.Ck, d.S, d.Bs, 1, off_k, perm_k, sort_scratch, st);
   if (rc != MUSE_OK) return rc;
   SummLayout L = summ_layout(d, dtype);
   char* base = (char*)summaries;
@@ -190,10 +224,12 @@ static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const i
   prof_mark("k_gather_rows", st);
   k_gather_rows<T><<<gg, 256, 0, st>>>(V, perm_k, d.N, D, Vp);
   MUSE_LAUNCH_OK();
+  if (counts != nullptr) {
+    prof_mark("k_bucket_sums", st);
+    k_bucket_sums<T, D><<<dim3(cdiv(d.Ck * d.S, 8), pk), 256, 0, st>>>(Kp, Vp, off_k, d.N, d.Ck * d.S, counts, ksum, vsum);
+    MUSE_LAUNCH_OK();
+  }
   if (d.SB == 0) return MUSE_OK;
-  Arena ar(ws);
-  int32_t* status = ar.take<int32_t>(sort_ws_elems(d.N, d.Ck * d.S) * (size_t)pk + 64) + sort_ws_elems(d.N, d.Ck * d.S) * (size_t)pk;
-  MUSE_CUDA_OK(cudaMemsetAsync(status, 0, 64 * sizeof(int32_t), st));     // 64 words after the sort scratch
   void* qsplit = ar.take<__nv_bfloat16>(2 * (size_t)d.B * d.Hq * d.Cq * d.D);   // split centroids for the tensor kernel
   rc = summarize_planes<T, D>(d, dtype, Kp, Vp, off_k, qbar, L, base, qsplit, status, st);
   if (rc != MUSE_OK || !d.dipole) return rc;
@@ -203,7 +239,7 @@ static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const i
 template <class T, int D>
 static int summarize_planes(const Dims& d, int dtype, const T* Kp, const T* Vp, const int32_t* off_k, const float* qbar,
                             const SummLayout& L, char* base, void* qsplit, int32_t* status, cudaStream_t st) {
-  if (summarize_tc_supported(d, dtype) && getenv("MUSE_SUMM_FWD_SIMT") == nullptr)
+  if (summarize_tc_supported(d, dtype) && !path_forced(kForceSummFwdSimt))
     return summarize_tc(d, Kp, Vp, off_k, qbar, summ_ptrs(L, base), qsplit, status, st);
   const size_t smem = (size_t)(kSumI * (D + 4) + kSumKC * (2 * D + 4) + kSumI * (kSumKC + 1)) * sizeof(float);
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
@@ -216,20 +252,22 @@ static int summarize_planes(const Dims& d, int dtype, const T* Kp, const T* Vp, 
 
 size_t summarize_ws_bytes(const Dims& d, int dtype) {
   Arena ar(nullptr);
-  ar.take<int32_t>((size_t)d.B * d.Hkv * sort_ws_elems(d.N, d.Ck * d.S) + 64);
+  ar.take<int32_t>(kStatusWords);
+  ar.take<int32_t>((size_t)d.B * d.Hkv * sort_ws_elems(d.N, d.Ck * d.S));
   ar.take<__nv_bfloat16>(2 * (size_t)d.B * d.Hq * d.Cq * d.D);
   return ar.used + dipole_ws_bytes(d, dtype);
 }
 
 int summarize(const Dims& d, int dtype, const void* K, const void* V, const int32_t* assign_k,
-              const float* qbar, int32_t* off_k, int32_t* perm_k, void* summaries, void* ws, cudaStream_t st) {
+              const float* qbar, int32_t* off_k, int32_t* perm_k, int32_t* counts, float* ksum, float* vsum,
+              void* summaries, void* ws, int32_t* status, cudaStream_t st) {
   if (dtype == MUSE_F32) {
-    if (d.D == 64) return summarize_t<float, 64>(d, dtype, (const float*)K, (const float*)V, assign_k, qbar, off_k, perm_k, summaries, ws, st);
-    return summarize_t<float, 128>(d, dtype, (const float*)K, (const float*)V, assign_k, qbar, off_k, perm_k, summaries, ws, st);
+    if (d.D == 64) return summarize_t<float, 64>(d, dtype, (const float*)K, (const float*)V, assign_k, qbar, off_k, perm_k, counts, ksum, vsum, summaries, ws, status, st);
+    return summarize_t<float, 128>(d, dtype, (const float*)K, (const float*)V, assign_k, qbar, off_k, perm_k, counts, ksum, vsum, summaries, ws, status, st);
   }
   typedef __nv_bfloat16 bf;
-  if (d.D == 64) return summarize_t<bf, 64>(d, dtype, (const bf*)K, (const bf*)V, assign_k, qbar, off_k, perm_k, summaries, ws, st);
-  return summarize_t<bf, 128>(d, dtype, (const bf*)K, (const bf*)V, assign_k, qbar, off_k, perm_k, summaries, ws, st);
+  if (d.D == 64) return summarize_t<bf, 64>(d, dtype, (const bf*)K, (const bf*)V, assign_k, qbar, off_k, perm_k, counts, ksum, vsum, summaries, ws, status, st);
+  return summarize_t<bf, 128>(d, dtype, (const bf*)K, (const bf*)V, assign_k, qbar, off_k, perm_k, counts, ksum, vsum, summaries, ws, status, st);
 }
 
 }  // namespace muse

@@ -259,7 +259,7 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
   tc::fence_before_sync();
   __syncthreads();
   if (warp == 0) tc::tmem_dealloc(tbase, 512);
-  if (!ok && tid == 0) atomicExch(status, 7);
+  if (!ok && tid == 0) report_status(status, 7);
 }
 
 bool summarize_tc_supported(const Dims& d, int dtype) { return dtype == MUSE_BF16 && d.D == st::D; }

@@ -23,11 +23,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait; false = gave up.  A correct kernel completes each wait within microseconds; the
-// limit only exists so that a logic error ends the kernel instead of hanging the GPU.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  for (int i = 0; i < (1 << 16); ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
+// limit (elapsed SM clocks, about half a second at 2 GHz by default) only exists so that a logic
+// error ends the kernel, which then reports through its status word, instead of hanging the GPU.
+constexpr uint32_t kWaitClocks = 1u << 30;
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, uint32_t limit_clocks = kWaitClocks) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const uint32_t t0 = (uint32_t)clock();
+  while (!mbar_try_wait(bar, parity))
+    if ((uint32_t)clock() - t0 > limit_clocks) return false;
+  return true;
 }
 
 // one arrival of the calling thread

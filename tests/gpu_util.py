@@ -73,3 +73,21 @@ class Case:
     def dev(self):
         d = self.w.dtype
         return to_dev(self.Q, d), to_dev(self.K, d), to_dev(self.V, d), to_dev(self.dO, d)
+
+
+class kernels_launched:
+    """Context manager: records the library's kernel names launched inside the block (through the
+    library's own per-kernel timing hook), so that a test can assert which path ran."""
+
+    def __enter__(self):
+        from paper_2509_10406_b200 import binding as mb
+        self.mb = mb
+        mb.muse_profile(True)
+        self.names = set()
+        return self
+
+    def __exit__(self, *exc):
+        torch.cuda.synchronize()
+        self.names = set(self.mb.muse_profile_report())
+        self.mb.muse_profile(False)
+        return False

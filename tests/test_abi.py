@@ -50,7 +50,7 @@ def test_invalid_parameters_are_rejected_on_the_host(mb, kw, code):
     args = dict(B=1, Hq=2, Hkv=2, N=1024, D=64, Cq=8, Ck=16, m=4)
     args.update(kw)
     p = mb.make_params(**args)
-    out = (ctypes.c_size_t * 5)()
+    out = (ctypes.c_size_t * 6)()
     assert mb.lib().muse_workspace_bytes(ctypes.byref(p), out) == code
     assert mb.lib().muse_strerror(code)
 
@@ -61,15 +61,23 @@ def test_null_and_small_workspace_are_rejected(mb):
     z = ctypes.c_void_p(0)
     assert L.muse_cluster(ctypes.byref(p), z, z, z, z, z, z, z, z, z, 0, z) == -1
     fake = ctypes.c_void_p(4096)      # aligned, never dereferenced: the size check comes first
-    assert L.muse_summarize(ctypes.byref(p), fake, fake, fake, fake, fake, fake, fake, fake, 16, z) == -3
+    assert L.muse_summarize(ctypes.byref(p), fake, fake, fake, fake, fake, fake, z, z, z, fake, fake, 16, z) == -3
+    # the three untilted outputs come together
+    assert L.muse_summarize(ctypes.byref(p), fake, fake, fake, fake, fake, fake, fake, z, z, fake, fake, 1 << 30, z) == -1
     assert L.muse_attn_fwd(ctypes.byref(p), fake, fake, fake, fake, fake, fake, fake, fake, z, fake, fake, z, fake, 16, z) == -3
     odd = ctypes.c_void_p(4100)
-    assert L.muse_summarize(ctypes.byref(p), odd, fake, fake, fake, fake, fake, fake, fake, 1 << 30, z) == -1
+    assert L.muse_summarize(ctypes.byref(p), odd, fake, fake, fake, fake, fake, z, z, z, fake, fake, 1 << 30, z) == -1
+    # backward without summaries needs the larger scratch
+    need = mb.muse_workspace_bytes(p)
+    assert need[5] == need[3] + need[4] + need[1]
+    a16 = [fake] * 9
+    assert L.muse_attn_bwd(ctypes.byref(p), fake, fake, fake, fake, fake, fake, fake, fake, fake, fake, z, fake,
+                           fake, fake, fake, fake, need[3], z) == -3
 
 
 def test_head_map(mb):
     p = mb.make_params(B=1, Hq=3, Hkv=2, N=1024, D=64, Cq=8, Ck=16, m=4, head_map=[0, 1, 1])
-    assert len(mb.muse_workspace_bytes(p)) == 5
+    assert len(mb.muse_workspace_bytes(p)) == 6
     p = mb.make_params(B=1, Hq=3, Hkv=2, N=1024, D=64, Cq=8, Ck=16, m=4, head_map=[0, 1, 2])
-    out = (ctypes.c_size_t * 5)()
+    out = (ctypes.c_size_t * 6)()
     assert mb.lib().muse_workspace_bytes(ctypes.byref(p), out) == -1

@@ -6,14 +6,21 @@ import pytest
 import torch
 
 from oracle import muse_oracle as orc
-from tests.gpu_util import Case, to_dev, to_np, tol, rel_err
+from tests.gpu_util import Case, to_dev, to_np, tol, rel_err, kernels_launched
 from tests.test_gpu_cluster import CASES
-from tests.test_gpu_forward import EDGE
+from tests.test_gpu_forward import EDGE, TC, TC_BWD_KERNELS
 
 pytestmark = pytest.mark.gpu
 
 
-def _backward_parity(w, gain, sel_mode=0, causal=True, agg_grad=True):
+def _backward_parity(w, gain, sel_mode=0, causal=True, agg_grad=True, expect_kernels=(), recompute=False):
+    with kernels_launched() as rec:
+        _backward_parity_run(w, gain, sel_mode, causal, agg_grad, recompute)
+    missing = set(expect_kernels) - rec.names
+    assert not missing, ("expected kernels did not run", missing, sorted(rec.names))
+
+
+def _backward_parity_run(w, gain, sel_mode=0, causal=True, agg_grad=True, recompute=False):
     from paper_2509_10406_b200 import binding as mb
     c = Case(w, gain=gain)
     qbar32 = c.qbar.astype(np.float32)
@@ -23,9 +30,14 @@ def _backward_parity(w, gain, sel_mode=0, causal=True, agg_grad=True):
     aq, qb = to_dev(c.a_q, "i"), to_dev(qbar32, "f32")
     mb.muse_summarize(p, K, V, to_dev(c.a_k, "i"), qb, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
     mb.muse_attn_fwd(p, Q, K, V, aq, qb, buf.off_k, buf.perm_k, buf.summaries, None, buf.O, buf.LSE, buf.sel, buf.ws)
-    mb.muse_attn_bwd(p, Q, K, V, buf.O, buf.LSE, dO, aq, qb, buf.off_k, buf.perm_k, buf.summaries, buf.sel,
-                     buf.dQ, buf.dK, buf.dV, buf.ws)
+    assert mb.muse_status(buf.ws) == 0
+    ws = buf.ws
+    if recompute:                                     # summaries = NULL: rebuilt inside the (larger) scratch
+        ws = torch.empty(buf.sizes[5], dtype=torch.uint8, device="cuda")
+    mb.muse_attn_bwd(p, Q, K, V, buf.O, buf.LSE, dO, aq, qb, buf.off_k, buf.perm_k, None if recompute else buf.summaries,
+                     buf.sel, buf.dQ, buf.dK, buf.dV, ws)
     torch.cuda.synchronize()
+    assert mb.muse_status(ws) == 0
     sel = to_np(buf.sel)[..., :w.m]
     dQ, dK, dV = to_np(buf.dQ), to_np(buf.dK), to_np(buf.dV)
     eQ, eK, eV = orc.layer_backward(c.Q.astype(np.float64), c.K.astype(np.float64), c.V.astype(np.float64),
@@ -60,6 +72,20 @@ def test_backward_per_query_cluster_selection():
 
 def test_backward_noncausal():
     _backward_parity(CASES["tiny"], 128.0, causal=False)
+
+
+@pytest.mark.parametrize("name", list(TC))
+@pytest.mark.parametrize("opt", ["default", "per_qcluster", "noncausal", "frozen_weights"])
+def test_backward_options_on_the_tensor_core_path(name, opt):
+    """Selection per query cluster, the non-causal mode and frozen aggregation weights on the shapes where
+    the tcgen05 far-field and key-side kernels run (the second case sums four query heads per kv head)."""
+    _backward_parity(TC[name], 128.0, sel_mode=1 if opt == "per_qcluster" else 0, causal=opt != "noncausal",
+                     agg_grad=opt != "frozen_weights", expect_kernels=TC_BWD_KERNELS)
+
+
+@pytest.mark.parametrize("name", ["tiny", "tc"])
+def test_backward_rebuilds_summaries_when_not_given(name):
+    _backward_parity(CASES["tiny"] if name == "tiny" else TC["tc"], 128.0, recompute=True)
 
 
 def test_backward_is_deterministic_for_dq():

@@ -7,7 +7,7 @@ import torch
 
 from oracle import muse_oracle as orc
 from paper_2509_10406_b200 import workloads as wl
-from tests.gpu_util import Case, to_dev, to_np, tol, rel_err
+from tests.gpu_util import Case, to_dev, to_np, tol, rel_err, kernels_launched
 from tests.test_gpu_cluster import CASES
 
 pytestmark = pytest.mark.gpu
@@ -15,6 +15,8 @@ pytestmark = pytest.mark.gpu
 EDGE = {
     "m0": CASES["gqa_bf16"].with_(B=1, Hq=2, Hkv=1, m=0),
     "one_block": CASES["tiny"].with_(S=1),
+    # one causal block in bf16: the block-diagonal tensor-core kernels alone, over the whole sequence
+    "one_block_bf16": CASES["d128"].with_(Hq=1, Hkv=1, N=2048, S=1, Cq=1, Ck=1, m=0),
     "one_qcluster": CASES["tiny"].with_(Cq=1, N=512),
     "tiny_blocks": CASES["tiny"].with_(N=64, Cq=2, Ck=8, m=8, components=4),
     "ragged_f32_d128": CASES["d128"].with_(dtype="f32", N=1000, Hq=1, Cq=8, Ck=24, m=3),
@@ -74,7 +76,24 @@ def test_summaries_match_oracle(name, gain):
             assert np.abs(e_beta[fin] - beta[b, h][fin]).max() <= 1e-4 * max(1.0, np.abs(e_beta[fin]).max())
 
 
-def _forward_parity(w, gain, sel_mode=0, causal=True):
+# bf16, D = 128, C_k a multiple of 128, C_q a multiple of 8: shapes at which every far-field, summary and
+# retrieval step runs its tcgen05 kernel; "tc_gqa4" has four query heads per kv head (the key-side group sum)
+TC = {
+    "tc": CASES["d128"].with_(name="tc", Hq=2, Hkv=1, N=4096, S=4, Cq=16, Ck=256, m=4),
+    "tc_gqa4": CASES["d128"].with_(name="tc_gqa4", Hq=4, Hkv=1, N=2048, S=4, Cq=8, Ck=128, m=4),
+}
+TC_FWD_KERNELS = {"k_summarize_tc", "k_far_fwd_tc", "k_local_fwd_tc"}
+TC_BWD_KERNELS = {"k_far_bwd_tc", "k_summ_bwd_tc"}
+
+
+def _forward_parity(w, gain, sel_mode=0, causal=True, expect_kernels=()):
+    with kernels_launched() as rec:
+        _forward_parity_run(w, gain, sel_mode, causal)
+    missing = set(expect_kernels) - rec.names
+    assert not missing, ("expected kernels did not run", missing, sorted(rec.names))
+
+
+def _forward_parity_run(w, gain, sel_mode=0, causal=True):
     mb, c, p, buf = _prep(w, gain, sel_mode=sel_mode, causal=causal)
     Q, K, V, _ = c.dev()
     _run_summaries(mb, c, p, buf, K, V)
@@ -84,6 +103,7 @@ def _forward_parity(w, gain, sel_mode=0, causal=True):
     mb.muse_attn_fwd(p, Q, K, V, to_dev(c.a_q, "i"), to_dev(c.qbar32, "f32"), buf.off_k, buf.perm_k, buf.summaries,
                      None, buf.O, buf.LSE, buf.sel, buf.ws)
     torch.cuda.synchronize()
+    assert mb.muse_status(buf.ws) == 0
     O_free, L_free, sel_gpu = to_np(buf.O), to_np(buf.LSE), to_np(buf.sel)[..., :w.m]
     stats = dict(sel_rows_differ=0, rows=0, err_forced_gpu_sel=0.0, err_forced_orc_sel=0.0)
     sel_orc = np.full((w.B, w.Hq, w.N, max(w.m, 1)), -1, np.int32)
@@ -135,6 +155,64 @@ def test_forward_per_query_cluster_selection():
 
 def test_forward_noncausal():
     _forward_parity(CASES["tiny"], 128.0, causal=False)
+
+
+@pytest.mark.parametrize("name", list(TC))
+@pytest.mark.parametrize("opt", ["default", "per_qcluster", "noncausal"])
+def test_forward_options_on_the_tensor_core_path(name, opt):
+    """Selection per query cluster and the non-causal (single block) mode on the shapes where the
+    tcgen05 kernels run, checked against the oracle like the default options."""
+    kern = TC_FWD_KERNELS - ({"k_local_fwd_tc"} if opt == "noncausal" else set())
+    _forward_parity(TC[name], 128.0, sel_mode=1 if opt == "per_qcluster" else 0, causal=opt != "noncausal",
+                    expect_kernels=kern)
+
+
+def test_untilted_bucket_statistics():
+    """counts, key sums and value sums per (cluster, block) bucket against their definition."""
+    for name in ("tiny", "gqa_bf16", "d128"):
+        mb, c, p, buf = _prep(CASES[name], 1.0)
+        w = c.w
+        Q, K, V, _ = c.dev()
+        dev = dict(device="cuda")
+        counts = torch.empty(w.B, w.Hkv, w.Ck, w.S, dtype=torch.int32, **dev)
+        ksum = torch.empty(w.B, w.Hkv, w.Ck, w.S, w.D, dtype=torch.float32, **dev)
+        vsum = torch.empty_like(ksum)
+        mb.muse_summarize(p, K, V, to_dev(c.a_k, "i"), to_dev(c.qbar32, "f32"), buf.off_k, buf.perm_k, buf.summaries, buf.ws,
+                          counts=counts, ksum=ksum, vsum=vsum)
+        torch.cuda.synchronize()
+        Bs = w.N // w.S
+        for b in range(w.B):
+            for g in range(w.Hkv):
+                key = c.a_k[b, g].astype(np.int64) * w.S + np.arange(w.N) // Bs
+                ec = np.bincount(key, minlength=w.Ck * w.S).reshape(w.Ck, w.S)
+                ek = np.zeros((w.Ck * w.S, w.D)); ev = np.zeros((w.Ck * w.S, w.D))
+                np.add.at(ek, key, c.K[b, g].astype(np.float64)); np.add.at(ev, key, c.V[b, g].astype(np.float64))
+                assert np.array_equal(to_np(counts)[b, g], ec)
+                assert rel_err(to_np(ksum)[b, g].reshape(-1, w.D), ek) <= 1e-5
+                assert rel_err(to_np(vsum)[b, g].reshape(-1, w.D), ev) <= 1e-5
+
+
+def test_out_of_range_selection_entries_count_as_none():
+    """sel_in entries outside [0, Ck) are treated as -1: same output as with -1 in their place, no CUDA error."""
+    mb, c, p, buf = _prep(TC["tc"], 128.0)
+    w = c.w
+    Q, K, V, _ = c.dev()
+    _run_summaries(mb, c, p, buf, K, V)
+    rng = np.random.default_rng(5)
+    sel = rng.integers(0, w.Ck, (w.B, w.Hq, w.N, w.m)).astype(np.int32)
+    sel[..., 1:] = -1                                  # one cluster per query, so that entries stay distinct
+    bad = sel.copy(); good = sel.copy()
+    rows = rng.choice(w.N, 64, replace=False)
+    bad[0, 0, rows, 1] = 0x7fffffff; bad[0, 1, rows, 2] = w.Ck; bad[0, 1, rows, 3] = -9
+    outs = []
+    for s_ in (good, bad):
+        mb.muse_attn_fwd(p, Q, K, V, to_dev(c.a_q, "i"), to_dev(c.qbar32, "f32"), buf.off_k, buf.perm_k, buf.summaries,
+                         to_dev(s_, "i"), buf.O, buf.LSE, buf.sel, buf.ws)
+        torch.cuda.synchronize()
+        assert mb.muse_status(buf.ws) == 0
+        outs.append((to_np(buf.O).copy(), to_np(buf.sel).copy()))
+    assert np.array_equal(outs[0][0], outs[1][0])
+    assert outs[1][1].max() < w.Ck and outs[1][1].min() >= -1
 
 
 @pytest.mark.parametrize("groups", [8, 2])

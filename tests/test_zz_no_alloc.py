@@ -31,10 +31,16 @@ def test_noalloc_cluster_matches_workspace_version_twice(name):
         out = mb.MuseBuffers(p, backward=False)
         for t in (out.assign_q, out.assign_k):
             t.fill_(-7)
-        before = torch.cuda.memory_allocated()
+        torch.cuda.synchronize()
+        # bytes the DRIVER reports free on the device: unlike torch's own counter, this would also see an
+        # allocation made inside the library.  The first call may load the library's device image (that is
+        # when its 32 MiB are reserved), so the comparison is made on the second call.
+        free_before = torch.cuda.mem_get_info()[0]
         mb.muse_cluster_noalloc(p, Q, K, iq, ik, out.assign_q, out.assign_k, out.qbar, out.kcent)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == before
+        if call == 1:
+            assert torch.cuda.mem_get_info()[0] >= free_before
+        assert mb.muse_cluster_noalloc_status() == 0
         got = [to_np(x) for x in (out.assign_q, out.assign_k, out.qbar, out.kcent)]
         assert np.array_equal(got[0], exp[0]) and np.array_equal(got[1], exp[1]), f"assignments differ on call {call}"
         assert np.abs(got[2] - exp[2]).max() <= 1e-6 * np.abs(exp[2]).max()
