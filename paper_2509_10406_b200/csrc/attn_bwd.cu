@@ -220,7 +220,7 @@ k_ret_bwd(Dims dm, const T* __restrict__ Q, const T* __restrict__ dO, const T* _
       const int vis_end = ok[pl + 1];
       if (c0 >= vis_end) continue;
       const int nk = min(kTile, vis_end - c0);
-      const int g0 = go[(size_t)pl * dm.Ck + j], g1 = go[(size_t)pl * dm.Ck + j + 1];
+      const int g0 = go[(size_t)j * dm.SB + pl], g1 = go[(size_t)j * dm.SB + pl + 1];
       for (int t0 = g0; t0 < g1; t0 += kTile) {
         const int nq = min(kTile, g1 - t0);
         __syncthreads();

@@ -259,7 +259,7 @@ k_ret_bwd_dq_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO
   const int j = blockIdx.x, pl = blockIdx.y / kRetSplitRows, sub = blockIdx.y % kRetSplitRows, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
-  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)pl * dm.Ck + j;
+  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)j * dm.SB + pl;
   const int g0 = go[0], g1 = go[1], ntiles = (g1 - g0 + kBM - 1) / kBM;
   if (sub >= ntiles) return;                          // this split has no pair tile
   const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
@@ -670,7 +670,7 @@ k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
   const int j = blockIdx.x, pl = blockIdx.y / kRetSplit, sub = blockIdx.y % kRetSplit, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
-  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)pl * dm.Ck + j;
+  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)j * dm.SB + pl;
   const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const int kbeg = ok[0], kvis = ok[pl + 1];
   const int g0 = go[0], g1 = go[1], ntiles = (g1 - g0 + kBN - 1) / kBN;
@@ -795,11 +795,11 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   const int j = blockIdx.x, sub = blockIdx.y, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
-  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + j;                // group of plane pl: go[pl * Ck], go[pl * Ck + 1]
+  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)j * dm.SB;   // group of plane pl: go[pl], go[pl + 1]
   const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const int k0 = ok[0], kall = ok[dm.SB];
   int ntiles_all = 0;
-  for (int pl = 0; pl < dm.SB; ++pl) ntiles_all += (go[(size_t)pl * dm.Ck + 1] - go[(size_t)pl * dm.Ck] + kBM - 1) / kBM;
+  for (int pl = 0; pl < dm.SB; ++pl) ntiles_all += (go[pl + 1] - go[pl] + kBM - 1) / kBM;
   // the tiles of the cluster are dealt round-robin to nsub CTAs (one for all but the most retrieved clusters)
   const int nsub = min(kFusedSplit, max(1, ntiles_all / kFusedTilesPerCta));
   if (ntiles_all == 0 || sub >= nsub) return;
@@ -842,13 +842,13 @@ k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   for (int kc0 = k0; kc0 < kall || kc0 == k0; kc0 += KC) {
     const bool first_sweep = kc0 == k0;
     auto plane_active = [&](int pl) {
-      const int g0 = go[(size_t)pl * dm.Ck], g1 = go[(size_t)pl * dm.Ck + 1];
+      const int g0 = go[pl], g1 = go[pl + 1];
       return g1 > g0;
     };
     auto first_from = [&](int pl) {
       Item it; it.pl = pl;
       while (it.pl < dm.SB && !plane_active(it.pl)) ++it.pl;
-      if (it.pl < dm.SB) { it.t0 = go[(size_t)it.pl * dm.Ck]; it.g1 = go[(size_t)it.pl * dm.Ck + 1]; } else { it.t0 = 0; it.g1 = 0; }
+      if (it.pl < dm.SB) { it.t0 = go[it.pl]; it.g1 = go[it.pl + 1]; } else { it.t0 = 0; it.g1 = 0; }
       return it;
     };
     auto next1 = [&](const Item& a) {

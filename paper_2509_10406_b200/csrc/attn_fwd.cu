@@ -22,7 +22,8 @@ __device__ __forceinline__ int query_plane(const Dims& d, int t) { return d.caus
 
 // ---------------------------------------------------------------------------------------------
 // Inverse index for retrieval (Section "Exact Retrieval and Local Attention"): for every
-// (plane, key cluster) the list of (query, slot) pairs that retrieve it.  Group key = plane * Ck + cluster.
+// (key cluster, plane) the list of (query, slot) pairs that retrieve it.  Group key = cluster * SB + plane,
+// so that the pairs of one cluster over all planes form one run, ordered by plane.
 // ---------------------------------------------------------------------------------------------
 // Thread e handles (slot = e / N, query = e % N): the lanes of a warp are consecutive queries,
 // which often retrieve the same cluster in the same slot, so equal keys are combined with a warp
@@ -35,7 +36,7 @@ __global__ void k_ret_count(Dims d, const int32_t* __restrict__ sel, int32_t* __
     const int t = (int)(e % d.N), k = (int)(e / d.N);
     const int c = sel[((size_t)pq * d.N + t) * d.m + k];
     const int pl = query_plane(d, t);
-    if (c >= 0 && c < d.Ck && pl >= 0) key = pl * d.Ck + c;      // entries outside [0, Ck) count as "none"
+    if (c >= 0 && c < d.Ck && pl >= 0) key = c * d.SB + pl;      // entries outside [0, Ck) count as "none"
   }
   const unsigned peers = __match_any_sync(0xffffffffu, key);
   const int lane = threadIdx.x & 31;
@@ -51,7 +52,7 @@ __global__ void k_ret_fill(Dims d, const int32_t* __restrict__ sel, int32_t* __r
     const int t = (int)(e % d.N), k = (int)(e / d.N);
     const int c = sel[((size_t)pq * d.N + t) * d.m + k];
     const int pl = query_plane(d, t);
-    if (c >= 0 && c < d.Ck && pl >= 0) { key = pl * d.Ck + c; pid = t * d.m + k; }
+    if (c >= 0 && c < d.Ck && pl >= 0) { key = c * d.SB + pl; pid = t * d.m + k; }
   }
   const unsigned peers = __match_any_sync(0xffffffffu, key);
   const int lane = threadIdx.x & 31, leader = __ffs(peers) - 1;
@@ -315,7 +316,7 @@ k_ret_fwd(Dims dm, const T* __restrict__ Q, const T* __restrict__ Kp, const T* _
   const int j = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
-  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)pl * dm.Ck + j;
+  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)j * dm.SB + pl;
   const int g0 = go[0], g1 = go[1];
   if (g0 >= g1) return;
   const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;

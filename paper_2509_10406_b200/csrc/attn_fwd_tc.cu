@@ -370,7 +370,7 @@ k_ret_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, c
   const int j = blockIdx.x, pl = blockIdx.y / kRetFwdSplit, sub = blockIdx.y % kRetFwdSplit, pq = blockIdx.z;
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int nkeys = dm.SB * dm.Ck;
-  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)pl * dm.Ck + j;
+  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)j * dm.SB + pl;
   const int g0 = go[0], g1 = go[1];
   if (g0 + sub * kTcM >= g1) return;                     // no pair tile for this split (before any TMEM allocation)
   const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
@@ -413,391 +413,6 @@ k_ret_fwd_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, c
   tc_teardown<D>(c, tid, status);
 }
 
-// ---- exact retrieval, cluster-resident version (D = 128) ---------------------------------------------
-// One CTA per (key cluster j, head): 128 of the cluster's keys and values stay in shared memory (two
-// chunks of 64) while the CTA walks the retrieving (query, slot) pairs of every plane in tiles of 128.
-// All logits of a tile come from one batch of MMAs, so the softmax needs no running rescale.  Eight
-// warps do the softmax and write the finished rows (staged, whole 256-byte rows); lane 0 of a ninth
-// warp issues every MMA, the logits of the next tile queued right behind the P V product of the
-// current one, whose output alternates between two accumulators so that nobody waits for it; three
-// more warps gather the Q rows one tile ahead, by asynchronous 16-byte copies into the other half of
-// a double buffer.  A cluster with more than 128 visible keys takes further sweeps, whose partial
-// results are merged into the stored rows by their log-sum-exp weights.
-constexpr int kRcThreads = 384, kRcCompute = 256, kRcIssuer = 256, kRcGather0 = 288, kRcGather = 96, kRcKeys = 128;
-constexpr int kRcSplit = 4, kRcTilesPerCta = 16;          // a cluster with many pair tiles is shared by up to 4 CTAs
-
-struct RcSmem {
-  static constexpr int D = 128;
-  static constexpr int kTile = kTcM * D * 2;               // 32 KB
-  static constexpr int q = 0, k = q + 2 * kTile, v = k + kRcKeys * D * 2, p = v + kRcKeys * D * 2,
-                       stage = p + 2 * kTcM * kTcN * 2, total = stage + kTile + 1024;
-  static constexpr uint32_t cS = 0, cO = 128, cols = 512;  // S (two chunks) | O of even tiles | O of odd tiles
-};
-
-__device__ __forceinline__ void rc_cp_async16(void* smem_dst, const void* src, bool valid) {
-  const int n = valid ? 16 : 0;                            // 0 source bytes: the 16 bytes are zero-filled
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(tc::smem_u32(smem_dst)), "l"(src), "r"(n) : "memory");
-}
-
-__global__ void __launch_bounds__(kRcThreads, 1)
-k_ret_fwd_cluster_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, const bf16* __restrict__ Vp,
-                     const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
-                     bf16* __restrict__ o_part, float* __restrict__ l_part, int* __restrict__ status) {
-  typedef RcSmem SM;
-  constexpr int D = SM::D;
-  extern __shared__ __align__(1024) unsigned char sm_raw[];
-  __shared__ uint64_t bar[2], bar_rows[2];                 // S ready / P V done / half b of the Q double buffer filled
-  __shared__ uint32_t tbase_s;
-  __shared__ int32_t pid_s[3][kTcM];                       // pair ids of the previous, the current and the next tile
-  __shared__ int32_t tok_s[2][kTcM];                       // tokens of the tile being gathered (alternating slots)
-  __shared__ float mx_s[2][kTcM], sum_s[2][kTcM], wold_s[kTcM], wnew_s[kTcM];
-  __shared__ int err_s;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = tid & 127, wg = (tid >> 7) & 1;
-  const bool cw = warp < 8, gw = warp >= 9;                // softmax warp / gather warp
-  const int j = blockIdx.x, sub = blockIdx.y, pq = blockIdx.z;
-  const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
-  const int nkeys = dm.SB * dm.Ck;
-  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + j;                // group of plane pl: go[pl * Ck], go[pl * Ck + 1]
-  const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
-  const int k0 = ok[0], kall = ok[dm.SB];
-  int ntiles_all = 0;
-  for (int pl = 0; pl < dm.SB; ++pl) ntiles_all += (go[(size_t)pl * dm.Ck + 1] - go[(size_t)pl * dm.Ck] + kTcM - 1) / kTcM;
-  // the tiles of the cluster are dealt round-robin to nsub CTAs (one for all but the most retrieved clusters)
-  const int nsub = min(kRcSplit, max(1, ntiles_all / kRcTilesPerCta));
-  if (ntiles_all == 0 || sub >= nsub) return;
-
-  unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
-  if (warp == 0) tc::tmem_alloc(&tbase_s, SM::cols);
-  if (tid == 0) {
-    tc::mbar_init(&bar[0], 1); tc::mbar_init(&bar[1], 1);
-    tc::mbar_init(&bar_rows[0], kRcGather); tc::mbar_init(&bar_rows[1], kRcGather);
-    tc::mbar_init_fence();
-    err_s = 0;
-  }
-  const bf16* Qb = Q + (size_t)pq * dm.N * D;
-  const bf16* Kb = Kp + (size_t)pk * dm.N * D;
-  const bf16* Vb = Vp + (size_t)pk * dm.N * D;
-  const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
-  tc::fence_async_smem();
-  tc::fence_before_sync();
-  __syncthreads();
-  tc::fence_after_sync();
-  const uint32_t tbase = tbase_s, tl = tbase + ((uint32_t)((warp & 3) * 32) << 16);
-  const uint32_t qa = tc::smem_u32(sm + SM::q), ka = tc::smem_u32(sm + SM::k), va = tc::smem_u32(sm + SM::v), pa = tc::smem_u32(sm + SM::p);
-  const float scale2 = dm.sigma * 1.4426950408889634f;
-  uint32_t ph0 = 0, ph1 = 0, ph_rows[2] = {0, 0};
-  bool ok_ = true;
-#ifdef MUSE_PHASE_CLOCKS
-  long long pc[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-  const long long t_in_ = clock64();
-#define RCLK(k) { long long n_ = clock64(); pc[k] += n_ - z_; z_ = n_; }
-#else
-#define RCLK(k)
-#endif
-  // Every warp walks the same sequence of tiles to the end, whatever happens (after a wait ran out the
-  // remaining waits are skipped), so the barriers below always see all their warps.
-  auto sync_cw_issuer = [&]() {                            // softmax warps and the issuing warp
-    if (!ok_) err_s = 1;
-    tc::fence_before_sync();
-    tc::named_bar_sync(2, kRcCompute + 32);
-    if (err_s) ok_ = false;
-  };
-  auto wait_rows = [&](int b) {
-    if (ok_ && !tc::mbar_wait(&bar_rows[b], ph_rows[b])) ok_ = false;
-    ph_rows[b] ^= 1;
-  };
-
-  struct Item { int pl, t0, g1; };
-  int kc0 = k0;                                             // first key of the current sweep
-  bool first_sweep = true;
-  auto first_from = [&](int pl) {
-    Item it; it.pl = pl; it.t0 = 0; it.g1 = 0;
-    while (it.pl < dm.SB && go[(size_t)it.pl * dm.Ck + 1] <= go[(size_t)it.pl * dm.Ck]) ++it.pl;
-    if (it.pl < dm.SB) { it.t0 = go[(size_t)it.pl * dm.Ck]; it.g1 = go[(size_t)it.pl * dm.Ck + 1]; }
-    return it;
-  };
-  auto next1 = [&](const Item& a) {
-    if (a.pl >= dm.SB) return a;
-    if (a.t0 + kTcM < a.g1) { Item it = a; it.t0 += kTcM; return it; }
-    return first_from(a.pl + 1);
-  };
-  auto skip = [&](Item a, int n) { for (int k = 0; k < n; ++k) a = next1(a); return a; };
-  // A tile belongs to the same CTA in every sweep (its position among ALL tiles of the cluster decides),
-  // because later sweeps add to the rows that the first one stored; from the second sweep on, the
-  // tiles of planes that see no key of the sweep are passed over.
-  auto live = [&](const Item& a) { return a.pl >= dm.SB || first_sweep || ok[a.pl + 1] > kc0; };
-  auto next_of = [&](Item a) { do { a = skip(a, nsub); } while (!live(a)); return a; };   // this CTA's next tile
-  auto first_of = [&]() { Item a = skip(first_from(0), sub); while (!live(a)) a = skip(a, nsub); return a; };
-  auto chunks_of = [&](const Item& a) {                                   // key chunks of this sweep that the tile's plane sees
-    return a.pl < dm.SB ? (min(kRcKeys, max(0, ok[a.pl + 1] - kc0)) + kTcN - 1) / kTcN : 0;
-  };
-  int pidreg = 0, tokreg = 0;
-  auto load_pids = [&](const Item& it) {
-    if (tid < kTcM) {
-      pidreg = (it.pl < dm.SB && it.t0 + tid < it.g1) ? __ldg(pr + it.t0 + tid) : 0;
-      tokreg = pidreg / dm.m;
-    }
-  };
-  // gather warps: Q rows of tile `it` (tokens tok[]) into half `b`; thread = 16-byte chunk g % 16 of rows
-  // g / 16 + 6 k, so that a warp copies two whole rows per instruction; rows past the end are zeros
-  auto gather_rows = [&](const Item& it, const int32_t* tok, int b) {
-    const int nq = min(kTcM, it.g1 - it.t0);
-    const int g = tid - kRcGather0, ck = g & 15;
-    unsigned char* qd = sm + SM::q + b * SM::kTile + (ck >> 3) * kTcM * 128;
-#pragma unroll 2
-    for (int r = g >> 4; r < kTcM; r += kRcGather / 16)
-      rc_cp_async16(qd + tc::sw128_off(r, ck & 7), Qb + (size_t)tok[r] * D + ck * 8, r < nq);
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    tc::fence_async_smem();                                 // the tensor cores read the rows through the async proxy
-    tc::mbar_arrive(&bar_rows[b]);
-  };
-  auto issue_s = [&](int b, int nch) {                      // issuer: logits of the tile whose rows are in half b
-    const uint32_t idesc = tc::idesc_bf16(kTcM, kTcN, 0, 0);
-    const uint32_t qab = qa + b * SM::kTile;
-    for (int ch = 0; ch < nch; ++ch) {
-#pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks)
-        tc::mma_bf16_ss(tbase + SM::cS + ch * kTcN, tc::smem_desc_sw128(qab + (ks / 4) * kTcM * 128 + (ks % 4) * 32, 16, 1024),
-                        tc::smem_desc_sw128(ka + ch * kTcN * D * 2 + (ks / 4) * kTcN * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
-    }
-    tc::mma_commit(&bar[0]);
-  };
-  // finished rows of the previous tile: normalised, bf16, staged, then stored 16 lanes per row (softmax warps)
-  int prev_nq = 0, prev_buf = 0, prev_o = 0;
-  float prev_inv = 0.f, prev_lse = 0.f;
-  bool pending = false, prev_first = true;
-  // The P V product of a tile is waited for before the next one can be issued (a parity wait must not fall
-  // two phases behind its barrier): by the next tile's softmax before it overwrites P, or by the deferred store.
-  bool pv_pending = false;
-  auto wait_pv = [&]() {
-    if (!pv_pending) return;                              // uniform over the CTA
-    if (ok_ && !tc::mbar_wait(&bar[1], ph1)) ok_ = false;
-    ph1 ^= 1;
-    tc::fence_after_sync();
-    pv_pending = false;
-  };
-  auto store_prev = [&]() {
-    if (!pending) return;                                 // uniform over the CTA
-    unsigned char* stg = sm + SM::stage;
-    wait_pv();
-#pragma unroll
-    for (int d0 = 0; d0 < D / 2; d0 += 32) {
-      float v[32];
-      tc::tmem_ld32(tl + SM::cO + prev_o * D + wg * (D / 2) + d0, v);
-#pragma unroll
-      for (int i = 0; i < 32; i += 8) {
-        uint32_t w[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          __nv_bfloat162 b2 = __floats2bfloat162_rn(v[i + 2 * e] * prev_inv, v[i + 2 * e + 1] * prev_inv);
-          w[e] = *reinterpret_cast<uint32_t*>(&b2);
-        }
-        const int ck = (wg * (D / 2) + d0 + i) >> 3;
-        *reinterpret_cast<uint4*>(stg + row * 256 + ((ck ^ (row & 15)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-      }
-    }
-    if (wg == 0 && row < prev_nq && ok_) {
-      float* lp = l_part + (size_t)pq * dm.N * dm.m + pid_s[prev_buf][row];
-      if (prev_first) {
-        *lp = prev_lse;
-      } else {
-        // merge with what earlier sweeps stored: weights exp(L_old - L), exp(L_new - L), L = log(e^L_old + e^L_new)
-        const float lo = *lp, ln = prev_lse, mxl = fmaxf(lo, ln);
-        const float eo = lo == -INFINITY ? 0.f : __expf(lo - mxl), en = ln == -INFINITY ? 0.f : __expf(ln - mxl);
-        const float tot = eo + en;
-        wold_s[row] = tot > 0.f ? eo / tot : 0.f;
-        wnew_s[row] = tot > 0.f ? en / tot : 0.f;
-        *lp = tot > 0.f ? mxl + __logf(tot) : -INFINITY;
-      }
-    }
-    tc::named_bar_sync(3, kRcCompute);
-    if (ok_) {
-      bf16* base = o_part + (size_t)pq * dm.N * dm.m * D;
-#pragma unroll
-      for (int k = 0; k < kTcM / 16; ++k) {
-        const int r = warp * 16 + 2 * k + (lane >> 4), ck = lane & 15;
-        if (r < prev_nq) {
-          uint4 val = *reinterpret_cast<const uint4*>(stg + r * 256 + ((ck ^ (r & 15)) << 4));
-          uint4* dst = reinterpret_cast<uint4*>(base + (size_t)pid_s[prev_buf][r] * D + ck * 8);
-          if (!prev_first) {
-            const uint4 old = *dst;
-            const float wo = wold_s[r], wn = wnew_s[r];
-            __nv_bfloat162* a2 = reinterpret_cast<__nv_bfloat162*>(&val);
-            const __nv_bfloat162* o2 = reinterpret_cast<const __nv_bfloat162*>(&old);
-#pragma unroll
-            for (int e = 0; e < 4; ++e)
-              a2[e] = __floats2bfloat162_rn(wn * __low2float(a2[e]) + wo * __low2float(o2[e]), wn * __high2float(a2[e]) + wo * __high2float(o2[e]));
-          }
-          *dst = val;
-        }
-      }
-    }
-    pending = false;
-  };
-
-  for (; kc0 < kall || first_sweep; kc0 += kRcKeys, first_sweep = false) {
-    __syncthreads();                                        // the previous sweep is done with the key / value tiles
-    // the cluster's keys (K-major for S = Q K^T) and values (MN-major for O = P V), two chunks of 64
-    if (cw) {
-      for (int ch = 0; ch < 2; ++ch) {
-        const int n = min(kTcN, max(0, kall - kc0 - ch * kTcN));
-        for (int e = tid; e < kTcN * (D / 8); e += kRcCompute) {
-          const int r = e / (D / 8), ck = e % (D / 8);
-          uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
-          if (r < n) {
-            a = reinterpret_cast<const uint4*>(Kb + (size_t)(kc0 + ch * kTcN + r) * D)[ck];
-            b = reinterpret_cast<const uint4*>(Vb + (size_t)(kc0 + ch * kTcN + r) * D)[ck];
-          }
-          const uint32_t off = ch * kTcN * D * 2 + (ck >> 3) * kTcN * 128 + tc::sw128_off(r, ck & 7);
-          *reinterpret_cast<uint4*>(sm + SM::k + off) = a;
-          *reinterpret_cast<uint4*>(sm + SM::v + off) = b;
-        }
-      }
-      tc::fence_async_smem();
-    }
-    Item cur = first_of(), nxt = next_of(cur), nn = next_of(nxt);
-    load_pids(cur);
-    if (tid < kTcM) { pid_s[0][tid] = pidreg; tok_s[0][tid] = tokreg; }
-    load_pids(nxt);
-    __syncthreads();
-    int buf = 0, qb = 0, tno = 0;                           // slot of the pair-id ring / half of the Q double buffer / tile count
-    if (gw && cur.pl < dm.SB) gather_rows(cur, tok_s[0], 0);
-    bool pre = false;                                       // the logits of the current tile are already issued
-    while (cur.pl < dm.SB) {
-#ifdef MUSE_PHASE_CLOCKS
-      long long z_ = clock64();
-#endif
-      const int nq = min(kTcM, cur.g1 - cur.t0);
-      const int vis = min(kRcKeys, max(0, ok[cur.pl + 1] - kc0));   // keys of this sweep that the plane sees
-      const int nch = (vis + kTcN - 1) / kTcN;
-      const int nbuf = buf == 2 ? 0 : buf + 1;
-      const int nch_next = chunks_of(nxt);
-      const bool pre_next = nch > 0 && nch_next > 0;        // this tile's last barrier also starts the next tile
-      if (tid < kTcM) { pid_s[nbuf][tid] = pidreg; tok_s[qb ^ 1][tid] = tokreg; }     // ids of the next tile
-      // ids of the next tile visible to the gather warps; the other half of the Q buffer was last read by the
-      // previous tile's logits, which the softmax warps have consumed
-      if (cw || gw) tc::named_bar_sync(1, kRcCompute + kRcGather);
-      if (gw) {
-        if (nxt.pl < dm.SB) gather_rows(nxt, tok_s[qb ^ 1], qb ^ 1);
-        cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf; qb ^= 1;
-        continue;
-      }
-      if (!pre) {
-        // first tile of the sweep, or the tile before had no key chunk: wait for this tile's rows here
-        if (cw) { wait_rows(qb); tc::fence_async_smem(); }
-        sync_cw_issuer();
-        if (tid == kRcIssuer && nch > 0) { tc::fence_after_sync(); issue_s(qb, nch); }
-      }
-      RCLK(0)
-      if (cw) load_pids(nn);
-      float M = -INFINITY, l = 0.f;
-      if (nch > 0) {
-        if (cw) {
-          if (ok_ && !tc::mbar_wait(&bar[0], ph0)) ok_ = false;
-          tc::fence_after_sync();
-          RCLK(1)
-          // softmax over up to 128 keys: each warpgroup takes 32 columns of every chunk; the two halves of a row
-          // meet through shared memory.  The logits are read from TMEM twice (row maximum, then probabilities)
-          // rather than kept in registers across the barrier.
-          float mx = -INFINITY;
-          for (int ch = 0; ch < nch; ++ch) {
-            float sv[32];
-            tc::tmem_ld32(tl + SM::cS + ch * kTcN + 32 * wg, sv);
-            const int visc = vis - ch * kTcN - 32 * wg;         // visible columns among these 32
-#pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, i < visc ? sv[i] : -INFINITY);
-          }
-          mx_s[wg][row] = mx * scale2;                          // (scale2 > 0)
-          RCLK(2)
-          tc::named_bar_sync(3, kRcCompute);
-          RCLK(3)
-          M = fmaxf(mx_s[0][row], mx_s[1][row]);
-          wait_pv();                                          // the previous P V product has read the P tiles
-          float rs = 0.f;
-          const float base = M == -INFINITY ? 0.f : M;
-          for (int ch = 0; ch < nch; ++ch) {
-            float sv[32];
-            tc::tmem_ld32(tl + SM::cS + ch * kTcN + 32 * wg, sv);
-            const int visc = vis - ch * kTcN - 32 * wg;
-            uint32_t pk[16];
-#pragma unroll
-            for (int i = 0; i < 32; i += 2) {
-              const float e0 = i < visc ? tc::fast_exp2(fmaf(sv[i], scale2, -base)) : 0.f;
-              const float e1 = i + 1 < visc ? tc::fast_exp2(fmaf(sv[i + 1], scale2, -base)) : 0.f;
-              __nv_bfloat162 b = __floats2bfloat162_rn(e0, e1);
-              rs += __low2float(b) + __high2float(b);          // the rounded values, as the P V product sees them
-              pk[i / 2] = *reinterpret_cast<uint32_t*>(&b);
-            }
-#pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4)
-              *reinterpret_cast<uint4*>(sm + SM::p + ch * kTcM * kTcN * 2 + tc::sw128_off(row, 4 * wg + c4)) =
-                  make_uint4(pk[c4 * 4], pk[c4 * 4 + 1], pk[c4 * 4 + 2], pk[c4 * 4 + 3]);
-          }
-          sum_s[wg][row] = rs;
-          RCLK(4)
-          if (pre_next) wait_rows(qb ^ 1);                    // the next tile's rows, for the logits issued below
-          tc::fence_async_smem();
-        }
-        ph0 ^= 1;
-        sync_cw_issuer();
-        RCLK(5)
-        if (tid == kRcIssuer) {
-          tc::fence_after_sync();
-          const uint32_t idesc = tc::idesc_bf16(kTcM, D, 0, 1);
-          for (int ch = 0; ch < nch; ++ch) {
-#pragma unroll
-            for (int ks = 0; ks < kTcN / 16; ++ks)
-              tc::mma_bf16_ss(tbase + SM::cO + (tno & 1) * D, tc::smem_desc_sw128(pa + ch * kTcM * kTcN * 2 + ks * 32, 16, 1024),
-                              tc::smem_desc_sw128(va + ch * kTcN * D * 2 + ks * 16 * 128, kTcN * 128, 1024), idesc, ch > 0 || ks > 0);
-          }
-          tc::mma_commit(&bar[1]);
-          if (pre_next) issue_s(qb ^ 1, nch_next);            // queued behind it: the next tile's logits
-        }
-        if (cw) l = sum_s[0][row] + sum_s[1][row];
-      }
-      if (cw) {
-        // The previous tile's rows leave now, while the tensor core works (the accumulators alternate).
-        store_prev();
-        RCLK(6)
-#ifdef MUSE_PHASE_CLOCKS
-        pc[7] += 1;
-#endif
-        pv_pending = nch > 0;                                 // this tile's product, waited for in the next tile
-        // what the deferred store needs: 1 / l and the log-sum-exp of the row (natural log)
-        prev_inv = l > 0.f ? 1.f / l : 0.f;
-        prev_lse = l > 0.f ? (M + log2f(l)) * 0.6931471805599453f : -INFINITY;
-        prev_nq = nq; prev_buf = buf; prev_o = tno & 1; pending = true; prev_first = first_sweep;
-        if (nch == 0) {
-          // nothing visible (possible with forced selections): rows of zeros, done here because the accumulator holds no data
-          if (row < nq && ok_) {
-            const size_t pid = (size_t)pq * dm.N * dm.m + pid_s[buf][row];
-            uint4* dst = reinterpret_cast<uint4*>(o_part + pid * D + wg * (D / 2));
-#pragma unroll
-            for (int i = 0; i < D / 16; ++i) dst[i] = make_uint4(0u, 0u, 0u, 0u);
-            if (wg == 0) l_part[pid] = -INFINITY;
-          }
-          pending = false;
-        }
-      }
-      pre = pre_next;
-      tc::fence_before_sync();
-      cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf; qb ^= 1; ++tno;
-    }
-    if (cw) store_prev();
-  }
-#ifdef MUSE_PHASE_CLOCKS
-  if (tid == 0 && pc[7] >= 12 && atomicCAS(status + 40, 0, 1) == 0) {
-    for (int k = 0; k < 8; ++k) status[41 + k] = (int)pc[k];
-    status[49] = (int)(clock64() - t_in_);
-  }
-#endif
-  tc::fence_before_sync();
-  __syncthreads();
-  if (warp == 0) tc::tmem_dealloc(tbase, SM::cols);
-  if (!ok_ && tid == 0) report_status(status, 1);
-}
-
 int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
 
 int local_fwd_tc(const Dims& d, const void* Q, const void* K, const void* V, float* o_loc, float* lse_loc, int* status,
@@ -820,18 +435,15 @@ int local_fwd_tc(const Dims& d, const void* Q, const void* K, const void* V, flo
   return MUSE_OK;
 }
 
+int ret_fwd_pairs_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
+                     const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st);
+
 int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
                const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st) {
   dim3 grid(d.Ck, d.SB * kRetFwdSplit, d.B * d.Hq);
   const int min_keys = 0;
-  if (d.D == 128 && !path_forced(kForceRetFwdStream)) {
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_cluster_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, RcSmem::total));
-    prof_mark("k_ret_fwd_cluster_tc", st);
-    k_ret_fwd_cluster_tc<<<dim3(d.Ck, kRcSplit, d.B * d.Hq), kRcThreads, RcSmem::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k,
-                                                                                 goff, pairs, (bf16*)o_part, l_part, status);
-    MUSE_LAUNCH_OK();
-    return MUSE_OK;
-  }
+  if (!path_forced(kForceRetFwdStream))
+    return ret_fwd_pairs_tc(d, Q, Kp, Vp, off_k, goff, pairs, o_part, l_part, status, st);
   prof_mark("k_ret_fwd_tc", st);
   if (d.D == 128) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdTcSmem<128>::total));

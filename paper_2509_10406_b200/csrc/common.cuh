@@ -110,7 +110,7 @@ __device__ __forceinline__ void report_status(int* status, int code) { atomicCAS
 // the tensor-core kernel (muse_test_force_paths; never set in production).
 enum ForcePath : unsigned {
   kForceSummFwdSimt = 1u, kForceFarSimt = 2u, kForceSummBwdSimt = 4u, kForceRetFwdStream = 8u,
-  kForceRetBwdSplit = 16u, kForceDipoleSimt = 32u, kForceRetFwdOld = 64u, kForceRetBwdOld = 128u
+  kForceRetBwdSplit = 16u, kForceDipoleSimt = 32u
 };
 bool path_forced(unsigned bit);
 
