@@ -77,7 +77,7 @@ def work_model(w: wl.Workload):
         "k_ret_bwd_dkdv_tc": ("tensor", heads * 8.0 * D * N * ret_keys),
         "k_ret_bwd_dq_tc": ("tensor", heads * 6.0 * D * N * ret_keys),
         "k_ret_fwd_pairs_tc": ("tensor", heads * 4.0 * D * N * ret_keys),
-        "k_ret_bwd_fused_tc": ("tensor", heads * 10.0 * D * N * ret_keys),    # S, dP, dQ, dK, dV from one gather
+        "k_ret_bwd_pairs_tc": ("tensor", heads * 10.0 * D * N * ret_keys),    # S, dP, dQ, dK, dV from one gather
         # merges and assembly
         "k_merge": ("hbm", heads * nd * (8 + e) + part + heads * N * m * 4),
         "k_final_dq": ("hbm", heads * nd * (4 + e) + part),

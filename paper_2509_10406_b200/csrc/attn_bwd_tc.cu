@@ -736,388 +736,6 @@ k_ret_bwd_dkdv_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ 
   bwd_teardown(c, SM::cols, tid, status);
 }
 
-// ================================================================================================
-// Fused retrieval backward (D = 128): one CTA per (key cluster j, head) walks every plane's group
-// of retrieving (query, slot) pairs in tiles of 128 pairs (pairs on the MMA M side), against the
-// cluster's keys in chunks of 64 (at most two chunks resident; longer clusters take another
-// sweep).  Per tile and key chunk:
-//   S = Q K^T, dP = dO V^T  ->  P = exp(sigma S - L), G = P (dP - delta)   (one thread per pair row)
-//   dQ   += G K                     [pairs][D]   written per pair as a bf16 row
-//   dV^T += dO^T P,  dK^T += Q^T G  [D][keys]    accumulated in TMEM over all tiles and planes
-// Eight warps do the arithmetic; lane 0 of a ninth warp issues every MMA, so that the first
-// products of the next chunk (or tile) queue behind the second batch of the current one; three
-// more warps gather.  The Q and dO rows of a tile are gathered once for all three products, one
-// tile ahead, by asynchronous 16-byte copies straight into the other half of a double buffer (the
-// load/store unit takes a few thousand cycles to accept a tile's 4096 copies: time the arithmetic
-// warps do not have); pair ids run two tiles ahead, across plane boundaries.  The CTA owns the cluster's keys for its head (or shares them with up
-// to three others): dK and dV leave as fire-and-forget adds, thread = output dim.
-// ================================================================================================
-constexpr int kFusedThreads = 384, kFusedCompute = 256, kFusedIssuer = 256, kFusedChunks = 2;
-constexpr int kFusedGather0 = 288, kFusedGather = 96;    // warps 9-11 gather rows; warps 0-8 meet at barrier 2, warps 0-7 and 9-11 at barrier 1
-constexpr int kFusedSplit = 4, kFusedTilesPerCta = 16;    // a cluster with many pair tiles is shared by up to 4 CTAs
-
-struct FusedSmem {
-  static constexpr int D = 128;
-  static constexpr int kTile = kBM * D * 2;                                // 32 KB
-  static constexpr int q = 0, dO = q + 2 * kTile, k = dO + 2 * kTile, v = k + kFusedChunks * kBN * D * 2,
-                       p = v + kFusedChunks * kBN * D * 2, g = p + kBM * kBN * 2,
-                       total = g + kBM * kBN * 2;   // 224 KB: no slack, the kernel checks the 1024-byte alignment of its base
-  static constexpr int stage = p;                                          // bf16 dQ rows on their way out: the P and G tiles together
-  static constexpr uint32_t cS = 0, cDP = 64, cDQ = 128, cDV = 256, cDK = 384, cols = 512;
-};
-
-__device__ __forceinline__ void cp_async16(void* smem_dst, const void* src, bool valid) {
-  const int n = valid ? 16 : 0;                                            // 0 source bytes: the 16 bytes are zero-filled
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(tc::smem_u32(smem_dst)), "l"(src), "r"(n) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
-
-__global__ void __launch_bounds__(kFusedThreads, 1)
-k_ret_bwd_fused_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO, const bf16* __restrict__ Kp,
-                   const bf16* __restrict__ Vp, const float* __restrict__ LSE, const float* __restrict__ delta,
-                   const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
-                   bf16* __restrict__ dq_part, float* __restrict__ dK_perm, float* __restrict__ dV_perm, int* __restrict__ status) {
-  typedef FusedSmem SM;
-#ifdef MUSE_PHASE_CLOCKS
-  const long long t_in_ = clock64();
-  long long t_l0_ = 0, t_l1_ = 0, t_pre_ = 0;
-#endif
-  constexpr int D = SM::D, KC = kFusedChunks * kBN;        // keys per sweep
-  extern __shared__ __align__(1024) unsigned char sm_raw[];
-  __shared__ uint64_t bar[2], bar_rows[2];                 // bar_rows[b]: half b of the row double buffer is filled
-  __shared__ uint32_t tbase_s;
-  __shared__ int32_t pid_s[3][kBM];                        // pair ids of the previous, the current and the next tile
-  __shared__ int32_t tok_s[2][kBM];                        // tokens of the tile being gathered (alternating slots)
-  __shared__ int err_s;
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, row = tid & 127, wg = (tid >> 7) & 1;
-  const bool cw = warp < 8, gw = warp >= 9;                // compute warp / gather warp
-  const int j = blockIdx.x, sub = blockIdx.y, pq = blockIdx.z;
-  const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
-  const int nkeys = dm.SB * dm.Ck;
-  const int32_t* go = goff + (size_t)pq * (nkeys + 1) + (size_t)j * dm.SB;   // group of plane pl: go[pl], go[pl + 1]
-  const int32_t* ok = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
-  const int k0 = ok[0], kall = ok[dm.SB];
-  int ntiles_all = 0;
-  for (int pl = 0; pl < dm.SB; ++pl) ntiles_all += (go[pl + 1] - go[pl] + kBM - 1) / kBM;
-  // the tiles of the cluster are dealt round-robin to nsub CTAs (one for all but the most retrieved clusters)
-  const int nsub = min(kFusedSplit, max(1, ntiles_all / kFusedTilesPerCta));
-  if (ntiles_all == 0 || sub >= nsub) return;
-  if (tc::smem_u32(sm_raw) & 1023u) {                      // the tiles fill the whole dynamic allocation: no room to realign
-    if (tid == 0) report_status(status, 2);
-    return;
-  }
-  if (tid == 0) { err_s = 0; tc::mbar_init(&bar_rows[0], kFusedGather); tc::mbar_init(&bar_rows[1], kFusedGather); }
-  uint32_t ph_rows[2] = {0, 0};
-  BwdCtx c;
-  bwd_setup(c, sm_raw, bar, &tbase_s, SM::cols, tid);
-#ifdef MUSE_PHASE_CLOCKS
-  t_pre_ = clock64();
-#endif
-  const bf16* Qb = Q + (size_t)pq * dm.N * D; const bf16* dOb = dO + (size_t)pq * dm.N * D;
-  const bf16* Kb = Kp + (size_t)pk * dm.N * D; const bf16* Vb = Vp + (size_t)pk * dm.N * D;
-  const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
-  // a wait that ran out on one thread ends the walk for all of them at the next barrier
-  auto sync_all = [&]() {                                  // arithmetic warps and the issuing warp
-    if (!c.ok) err_s = 1;
-    tc::fence_before_sync();
-    tc::named_bar_sync(2, kFusedCompute + 32);
-    if (err_s) c.ok = false;
-  };
-  // Every warp walks the same sequence of tiles to the end, whatever happens (after a wait ran out the
-  // remaining waits are skipped): the barriers below always see all their warps.
-  auto wait_rows = [&](int b) {
-    if (c.ok && !tc::mbar_wait(&bar_rows[b], ph_rows[b])) c.ok = false;
-    ph_rows[b] ^= 1;
-  };
-  const uint32_t qa = tc::smem_u32(c.sm + SM::q), da = tc::smem_u32(c.sm + SM::dO), ka = tc::smem_u32(c.sm + SM::k),
-                 va = tc::smem_u32(c.sm + SM::v), pa = tc::smem_u32(c.sm + SM::p), ga = tc::smem_u32(c.sm + SM::g);
-  const uint32_t tl = c.tbase + ((uint32_t)((warp & 3) * 32) << 16);
-  const float scale2 = dm.sigma * kLog2e;
-
-  // work items: (plane, first pair of the tile).  A tile belongs to the same CTA in every sweep (its position
-  // among ALL tiles of the cluster decides), because later sweeps add to the dQ rows that the first one stored;
-  // from the second sweep on, the tiles of planes that see no key of the sweep are passed over.
-  struct Item { int pl, t0, g1; };
-  for (int kc0 = k0; kc0 < kall || kc0 == k0; kc0 += KC) {
-    const bool first_sweep = kc0 == k0;
-    auto plane_active = [&](int pl) {
-      const int g0 = go[pl], g1 = go[pl + 1];
-      return g1 > g0;
-    };
-    auto first_from = [&](int pl) {
-      Item it; it.pl = pl;
-      while (it.pl < dm.SB && !plane_active(it.pl)) ++it.pl;
-      if (it.pl < dm.SB) { it.t0 = go[it.pl]; it.g1 = go[it.pl + 1]; } else { it.t0 = 0; it.g1 = 0; }
-      return it;
-    };
-    auto next1 = [&](const Item& a) {
-      if (a.pl >= dm.SB) return a;
-      if (a.t0 + kBM < a.g1) { Item it = a; it.t0 += kBM; return it; }
-      return first_from(a.pl + 1);
-    };
-    auto skip = [&](Item a, int n) { for (int k = 0; k < n; ++k) a = next1(a); return a; };
-    auto live = [&](const Item& a) { return a.pl >= dm.SB || first_sweep || ok[a.pl + 1] > kc0; };
-    auto next_of = [&](Item a) { do { a = skip(a, nsub); } while (!live(a)); return a; };   // this CTA's next tile
-    auto first_of = [&]() { Item a = skip(first_from(0), sub); while (!live(a)) a = skip(a, nsub); return a; };
-    auto chunks_of = [&](const Item& a) {                                 // key chunks of this sweep that the tile's plane sees
-      return a.pl < dm.SB ? (min(KC, max(0, ok[a.pl + 1] - kc0)) + kBN - 1) / kBN : 0;
-    };
-    // key / value chunks of this sweep
-    __syncthreads();
-    const int nkc = min(KC, kall - kc0);                    // keys of the sweep that any plane sees
-    if (cw) {
-#pragma unroll
-      for (int ch = 0; ch < kFusedChunks; ++ch) {
-        const int n = min(kBN, max(0, nkc - ch * kBN));
-        fill_tile<D, kBN, kFusedCompute>(c.sm + SM::k + ch * kBN * D * 2, n, [&](int r) { return Kb + (size_t)(kc0 + ch * kBN + r) * D; }, tid);
-        fill_tile<D, kBN, kFusedCompute>(c.sm + SM::v + ch * kBN * D * 2, n, [&](int r) { return Vb + (size_t)(kc0 + ch * kBN + r) * D; }, tid);
-      }
-    }
-    bool started[kFusedChunks] = {false, false};            // dV^T / dK^T of chunk ch hold something
-
-    float Lreg = 0.f, dreg = 0.f;
-    int pidreg = 0, tokreg = 0;
-    auto load_pids = [&](const Item& it) {
-      if (tid < kBM) {
-        pidreg = (it.pl < dm.SB && it.t0 + tid < it.g1) ? __ldg(pr + it.t0 + tid) : 0;
-        tokreg = pidreg / dm.m;
-      }
-    };
-    // gather warps: rows of tile `it` (tokens tok[]) into half `b` of the double buffer; thread = 16-byte chunk
-    // g % 16 of rows g / 16 + 6 k, so that a warp copies two whole rows per instruction; rows past the end are zeros
-    auto gather_rows = [&](const Item& it, const int32_t* tok, int b) {
-      const int nq = min(kBM, it.g1 - it.t0);
-      const int g = tid - kFusedGather0, ck = g & 15;
-      unsigned char* qd = c.sm + SM::q + b * SM::kTile + (ck >> 3) * kBM * 128;
-      unsigned char* od = c.sm + SM::dO + b * SM::kTile + (ck >> 3) * kBM * 128;
-#pragma unroll 2
-      for (int r = g >> 4; r < kBM; r += kFusedGather / 16) {
-        const size_t at = (size_t)tok[r] * D + ck * 8;
-        cp_async16(qd + tc::sw128_off(r, ck & 7), Qb + at, r < nq);
-        cp_async16(od + tc::sw128_off(r, ck & 7), dOb + at, r < nq);
-      }
-      cp_async_commit();
-      cp_async_wait_all();
-      tc::fence_async_smem();                               // the tensor cores read the rows through the async proxy
-      tc::mbar_arrive(&bar_rows[b]);
-    };
-    // arithmetic warps: L and delta of the tile's rows, one tile ahead
-    auto load_row_scalars = [&](const Item& it, const int32_t* tok) {
-      const int nq = min(kBM, it.g1 - it.t0);
-      const size_t tt = (size_t)pq * dm.N + tok[row];
-      Lreg = row < nq ? LSE[tt] * kLog2e : 0.f;
-      dreg = row < nq ? delta[tt] : 0.f;
-    };
-    auto issue_first = [&](int b, int ch) {                                // issuer: S = Q K^T and dP = dO V^T for key chunk ch
-      const uint32_t kac = ka + ch * kBN * D * 2, vac = va + ch * kBN * D * 2, qab = qa + b * SM::kTile, dab = da + b * SM::kTile;
-      const uint32_t idesc = tc::idesc_bf16(kBM, kBN, 0, 0);
-#pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase + SM::cS, desc_k<kBM>(qab, ks), desc_k<kBN>(kac, ks), idesc, ks > 0);
-#pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks) tc::mma_bf16_ss(c.tbase + SM::cDP, desc_k<kBM>(dab, ks), desc_k<kBN>(vac, ks), idesc, ks > 0);
-      tc::mma_commit(&c.bar[0]);
-    };
-    Item cur = first_of(), nxt = next_of(cur), nn = next_of(nxt);
-    load_pids(cur);
-    if (tid < kBM) { pid_s[0][tid] = pidreg; tok_s[0][tid] = tokreg; }
-    load_pids(nxt);
-    __syncthreads();
-    int buf = 0, qb = 0;                                     // slot of the pair-id ring / half of the row double buffer
-    if (cur.pl < dm.SB) {
-      if (gw) gather_rows(cur, tok_s[0], 0);
-      if (cw) load_row_scalars(cur, tok_s[0]);
-    }
-    // The dQ rows of a tile are written while the first products of the NEXT tile run on the tensor cores
-    // (the accumulator columns are only overwritten by that tile's second batch of MMAs).
-    int prev_nq = 0, prev_nch = -1, prev_buf = 0;          // prev_nch < 0: nothing pending
-    auto store_dq = [&]() {                                 // compute warps only
-      if (prev_nch < 0) return;                                         // uniform over the CTA
-      const uint32_t tq = tl + SM::cDQ + wg * (D / 2);
-      bf16* base = dq_part + (size_t)pq * dm.N * dm.m * D;
-      // bf16 rows go through a staging tile (thread = row, 16-byte chunks XOR-swizzled) so that they
-      // leave as whole 256-byte rows, 16 lanes per row: a row-per-thread store would touch 32 lines per
-      // instruction.  Later sweeps (clusters with more keys than one sweep holds) add to the stored rows.
-      unsigned char* stg = c.sm + SM::stage;
-#pragma unroll
-      for (int d0 = 0; d0 < D / 2; d0 += 32) {
-        float v[32];
-        if (prev_nch > 0) tc::tmem_ld32(tq + d0, v);
-#pragma unroll
-        for (int i = 0; i < 32; i += 8) {
-          uint32_t w[4];
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            __nv_bfloat162 b2 = prev_nch > 0 ? __floats2bfloat162_rn(v[i + 2 * e], v[i + 2 * e + 1]) : __floats2bfloat162_rn(0.f, 0.f);
-            w[e] = *reinterpret_cast<uint32_t*>(&b2);
-          }
-          const int ck = (wg * (D / 2) + d0 + i) >> 3;
-          *reinterpret_cast<uint4*>(stg + row * 256 + ((ck ^ (row & 15)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-        }
-      }
-      tc::named_bar_sync(3, kFusedCompute);
-      if (c.ok) {
-#pragma unroll
-        for (int k = 0; k < kBM / 16; ++k) {                            // 8 warps x 8 steps x 2 rows
-          const int r = warp * 16 + 2 * k + (lane >> 4), ck = lane & 15;
-          if (r < prev_nq) {
-            uint4 val = *reinterpret_cast<const uint4*>(stg + r * 256 + ((ck ^ (r & 15)) << 4));
-            uint4* dst = reinterpret_cast<uint4*>(base + (size_t)pid_s[prev_buf][r] * D + ck * 8);
-            if (!first_sweep) {
-              const uint4 old = *dst;
-              __nv_bfloat162* a2 = reinterpret_cast<__nv_bfloat162*>(&val);
-              const __nv_bfloat162* o2 = reinterpret_cast<const __nv_bfloat162*>(&old);
-#pragma unroll
-              for (int e = 0; e < 4; ++e) a2[e] = __floats2bfloat162_rn(__low2float(a2[e]) + __low2float(o2[e]), __high2float(a2[e]) + __high2float(o2[e]));
-            }
-            *dst = val;
-          }
-        }
-      }
-      tc::named_bar_sync(3, kFusedCompute);                             // the staging space is the P / G tiles
-      prev_nch = -1;
-    };
-#ifdef MUSE_PHASE_CLOCKS
-    t_l0_ = clock64();
-#endif
-    bool pre = false;                                       // the first products of the current tile are already issued
-    while (cur.pl < dm.SB) {
-#ifdef MUSE_PHASE_CLOCKS
-      long long z_ = clock64();
-#define ZCLK(k) { long long n_ = clock64(); c.pc[k] += n_ - z_; z_ = n_; }
-#else
-#define ZCLK(k)
-#endif
-      const int nq = min(kBM, cur.g1 - cur.t0);
-      const int vis = min(KC, max(0, ok[cur.pl + 1] - kc0));            // keys of this sweep that the plane sees
-      const int nch = (vis + kBN - 1) / kBN;
-      const int nbuf = buf == 2 ? 0 : buf + 1;
-      const bool pre_next = nch > 0 && chunks_of(nxt) > 0;              // this tile's last barrier also starts the next tile
-      if (tid < kBM) { pid_s[nbuf][tid] = pidreg; tok_s[qb ^ 1][tid] = tokreg; }   // ids of the next tile
-      const float L2 = Lreg, dl = dreg;
-      // ids of the next tile visible to the gather warps; the other half of the row buffer was last read by the
-      // previous tile's MMAs, which the arithmetic warps have waited for
-      if (cw || gw) tc::named_bar_sync(1, kFusedCompute + kFusedGather);
-      if (gw) {
-        if (nxt.pl < dm.SB) gather_rows(nxt, tok_s[qb ^ 1], qb ^ 1);
-        cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf; qb ^= 1;
-        continue;
-      }
-      if (!pre) {
-        // first tile of the sweep, or the tile before had no key chunk: wait for this tile's rows here
-        if (cw) { wait_rows(qb); tc::fence_async_smem(); }
-        sync_all();
-        if (tid == kFusedIssuer && nch > 0) { tc::fence_after_sync(); issue_first(qb, 0); }
-      }
-      ZCLK(0)
-      if (cw) {
-        if (nxt.pl < dm.SB) load_row_scalars(nxt, tok_s[qb ^ 1]);
-        load_pids(nn);
-        store_dq();                                                     // previous tile's rows leave while the first products run
-      }
-      ZCLK(1)
-      for (int ch = 0; ch < nch; ++ch) {
-        const bool last = ch + 1 == nch;
-        if (cw) {
-          if (c.ok && !tc::mbar_wait(&c.bar[0], c.ph0)) c.ok = false;
-          tc::fence_after_sync();
-          ZCLK(2)
-          const int visc = min(kBN, vis - ch * kBN);
-          float sv[32], dp[32], pv[32], gv[32];
-          tc::tmem_ld32(tl + SM::cS + 32 * wg, sv);
-          tc::tmem_ld32(tl + SM::cDP + 32 * wg, dp);
-#pragma unroll
-          for (int i = 0; i < 32; ++i) {
-            const float e = tc::fast_exp2(sv[i] * scale2 - L2);
-            pv[i] = (row < nq && 32 * wg + i < visc) ? e : 0.f;
-            gv[i] = pv[i] * (dp[i] - dl) * dm.sigma;                    // (sigma rides on G: dQ and dK come out scaled)
-          }
-          if (ch > 0) {                                                 // the previous chunk's MMAs have read P / G
-            if (c.ok && !tc::mbar_wait(&c.bar[1], c.ph1)) c.ok = false;
-            c.ph1 ^= 1;
-          }
-          store_row32(c.sm + SM::p, row, wg, pv);
-          store_row32(c.sm + SM::g, row, wg, gv);
-          ZCLK(3)
-          if (last && pre_next) wait_rows(qb ^ 1);                      // the next tile's rows, for the products issued below
-          tc::fence_async_smem();
-          ZCLK(4)
-        }
-        c.ph0 ^= 1;
-        sync_all();
-        ZCLK(5)
-        if (tid == kFusedIssuer) {
-          tc::fence_after_sync();
-          const uint32_t kac = ka + ch * kBN * D * 2, qab = qa + qb * SM::kTile, dab = da + qb * SM::kTile;
-          const uint32_t id_dq = tc::idesc_bf16(kBM, D, 0, 1);          // A = G (contraction over keys), B = key rows MN-major
-          const uint32_t id_t = tc::idesc_bf16(D, kBN, 1, 1);           // A = dO / Q tile and B = P / G tile, both contracted over pairs
-#pragma unroll
-          for (int ks = 0; ks < kBN / 16; ++ks)
-            tc::mma_bf16_ss(c.tbase + SM::cDQ, tc::smem_desc_sw128(ga + ks * 32, 16, 1024), desc_mn<kBN>(kac, ks), id_dq, ch > 0 || ks > 0);
-#pragma unroll
-          for (int ks = 0; ks < kBM / 16; ++ks)
-            tc::mma_bf16_ss(c.tbase + SM::cDV + ch * kBN, desc_mn<kBM>(dab, ks), tc::smem_desc_sw128(pa + ks * 16 * 128, kBM * 128, 1024), id_t,
-                            started[ch] || ks > 0);
-#pragma unroll
-          for (int ks = 0; ks < kBM / 16; ++ks)
-            tc::mma_bf16_ss(c.tbase + SM::cDK + ch * kBN, desc_mn<kBM>(qab, ks), tc::smem_desc_sw128(ga + ks * 16 * 128, kBM * 128, 1024), id_t,
-                            started[ch] || ks > 0);
-          tc::mma_commit(&c.bar[1]);
-          // queued behind them: the first products of the next chunk, or of the next tile
-          if (!last) issue_first(qb, ch + 1);
-          else if (pre_next) issue_first(qb ^ 1, 0);
-        }
-        started[ch] = true;
-      }
-      if (cw && nch > 0) {                                              // the last chunk's MMAs: dQ complete, both halves of the buffers free
-        if (c.ok && !tc::mbar_wait(&c.bar[1], c.ph1)) c.ok = false;
-        c.ph1 ^= 1;
-        tc::fence_after_sync();
-      }
-      ZCLK(5)
-#ifdef MUSE_PHASE_CLOCKS
-      c.pc[7] += 1;
-#endif
-      pre = pre_next;
-      prev_nq = nq; prev_nch = nch; prev_buf = buf;
-      tc::fence_before_sync();
-      cur = nxt; nxt = nn; nn = next_of(nn); buf = nbuf; qb ^= 1;
-    }
-#ifdef MUSE_PHASE_CLOCKS
-    t_l1_ = clock64();
-#endif
-    if (cw) {
-      store_dq();
-      // dV (warpgroup 0) and dK (warpgroup 1) of this sweep's keys: thread = output dim, one key per column
-#pragma unroll
-      for (int ch = 0; ch < kFusedChunks; ++ch) {
-        if (!started[ch]) continue;                                     // uniform over the CTA
-        const int n = min(kBN, nkc - ch * kBN);
-        float* dst = (wg == 0 ? dV_perm : dK_perm) + ((size_t)pq * dm.N + kc0 + ch * kBN) * D + row;
-#pragma unroll
-        for (int u0 = 0; u0 < kBN; u0 += 32) {
-          float v[32];
-          tc::tmem_ld32(tl + (wg == 0 ? SM::cDV : SM::cDK) + ch * kBN + u0, v);
-          if (c.ok) {
-#pragma unroll
-            for (int u = 0; u < 32; ++u)
-              if (u0 + u < n) atomicAdd(dst + (size_t)(u0 + u) * D, v[u]);       // (result unused: no round trip)
-          }
-        }
-      }
-    }
-    tc::fence_before_sync();
-  }
-#ifdef MUSE_PHASE_CLOCKS
-  if (tid == 0 && c.pc[7] >= 12 && atomicCAS(status + 40, 0, 1) == 0)
-  {
-    for (int k = 0; k < 8; ++k) status[41 + k] = (int)c.pc[k];
-    status[49] = (int)(t_pre_ - t_in_); status[50] = (int)(t_l0_ - t_in_); status[51] = (int)(t_l1_ - t_l0_); status[52] = (int)(clock64() - t_l1_);
-  }
-#endif
-  bwd_teardown(c, SM::cols, tid, status);
-}
-
 // ---- launchers ------------------------------------------------------------------------------------
 #define MUSE_TC_LAUNCH(KERNEL, SMEM, NT, GRID, ...)                                                                  \
   do {                                                                                                            \
@@ -1149,18 +767,16 @@ int local_bwd_tc(const Dims& d, const void* Q, const void* K, const void* V, con
   return MUSE_OK;
 }
 
+int ret_bwd_pairs_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, const void* Vp, const float* LSE,
+                     const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, void* dq_part,
+                     float* dK_perm, float* dV_perm, int* status, cudaStream_t st);
+
 int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, const void* Vp, const float* LSE,
                const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, void* dq_part,
                float* dK_perm, float* dV_perm, int* status, cudaStream_t st) {
   const int pq = d.B * d.Hq;
-  if (d.D == 128 && !path_forced(kForceRetBwdSplit)) {
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_bwd_fused_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, FusedSmem::total));
-    prof_mark("k_ret_bwd_fused_tc", st);
-    k_ret_bwd_fused_tc<<<dim3(d.Ck, kFusedSplit, pq), kFusedThreads, FusedSmem::total, st>>>(d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp, (const bf16*)Vp,
-                                                                               LSE, delta, off_k, goff, pairs, (bf16*)dq_part, dK_perm, dV_perm, status);
-    MUSE_LAUNCH_OK();
-    return MUSE_OK;
-  }
+  if (d.D == 128 && !path_forced(kForceRetBwdSplit))
+    return ret_bwd_pairs_tc(d, Q, dO, Kp, Vp, LSE, delta, off_k, goff, pairs, dq_part, dK_perm, dV_perm, status, st);
   prof_mark("k_ret_bwd_dkdv_tc", st);
   MUSE_TC_LAUNCH(k_ret_bwd_dkdv_tc, KeysSmem, kKeysThreads, dim3(d.Ck, d.SB * kRetSplit, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,
                  (const bf16*)Vp, LSE, delta, off_k, goff, pairs, dK_perm, dV_perm, status);

@@ -10,10 +10,12 @@
 //                           normalised and stored as a bf16 partial row with its log-sum-exp (the
 //                           merge kernel combines a query's slots)
 // Warp roles: warps 0-3 softmax and read-out (thread = pair row), lane 0 of warp 4 issues the MMAs,
-// warps 5-6 gather the Q rows of the next tile (16-byte asynchronous copies; the load/store unit
-// accepts them slowly, which is why no arithmetic warp issues them) as soon as the first product has
-// released the single Q buffer.  The CTA is deliberately small (96 KB of shared memory, 256 TMEM
-// columns, 224 threads) so that two of them share an SM and fill each other's waits.
+// warps 5-6 gather the Q rows of the next tile as soon as the first product has released the single Q
+// buffer (16-byte asynchronous copies; an SM's load/store unit moves such scattered 256-byte rows at
+// about 25 bytes per clock at best, so no arithmetic warp should spend its time issuing them; more
+// gather warps were slower: their copies crowd out the row warps' stores).  The CTA is deliberately
+// small (96 KB of shared memory, 256 TMEM columns, 224 threads) so that two of them share an SM and
+// fill each other's waits.
 // Clusters with more than 128 visible keys take further sweeps over the tiles that see them; a later
 // sweep merges its partial result into the stored row by log-sum-exp weights.
 #include <cuda.h>
@@ -25,7 +27,7 @@ namespace muse {
 typedef __nv_bfloat16 bf16;
 
 namespace rf {
-constexpr int kRowThreads = 128, kIssuerWarp = 4, kGather0 = 160, kGather = 64, kThreads = 224;
+constexpr int kRowThreads = 128, kIssuerWarp = 4, kGather0 = 160, kGather = 64, kThreads = kGather0 + kGather;
 constexpr int kPairs = 128, kKeys = 128;
 constexpr int kSplit = 4, kTilesPerCta = 8;                // a cluster with many pair tiles is shared by up to 4 CTAs
 constexpr int kOkCache = 72;                               // bucket offsets of the cluster kept in shared memory (S + 1 <= 72)
@@ -41,14 +43,6 @@ struct Bars { uint64_t q_full, q_empty, s_done, p_ready, o_done, o_free; };
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* src, bool valid) {
   const int n = valid ? 16 : 0;                            // 0 source bytes: the 16 bytes are zero-filled
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(tc::smem_u32(smem_dst)), "l"(src), "r"(n) : "memory");
-}
-__device__ __forceinline__ void st_global_32B(void* dst, const uint32_t (&w)[8]) {
-  asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]),
-               "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]) : "memory");
-}
-__device__ __forceinline__ void ld_global_32B(const void* src, uint32_t (&w)[8]) {
-  asm volatile("ld.global.v8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];" : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]),
-               "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]) : "l"(src) : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]: A is a 128-row bf16 matrix in tensor memory, two K-elements per 32-bit column
 __device__ __forceinline__ void mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
@@ -247,7 +241,7 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
             for (int c = 0; c < 2; ++c) {                            // 16 columns = 32 bytes per store
               uint32_t w[8];
               if (!first) {
-                ld_global_32B(orow + d0 + 16 * c, w);
+                tc::ld_global_32B(orow + d0 + 16 * c, w);
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                   const __nv_bfloat162 o2 = *reinterpret_cast<const __nv_bfloat162*>(&w[e]);
@@ -262,7 +256,7 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
                   w[e] = *reinterpret_cast<uint32_t*>(&b2);
                 }
               }
-              st_global_32B(orow + d0 + 16 * c, w);
+              tc::st_global_32B(orow + d0 + 16 * c, w);
             }
           }
         }
@@ -316,22 +310,23 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       const int g = tid - kGather0, ck = g % CPR;
       constexpr int RPP = kGather / CPR;                   // rows per pass
       unsigned char* qd = sm + SM::q + (ck >> 3) * kPairs * 128;
-      auto tile_pids = [&](int t, int& a, int& b, int& last) {      // ids of rows g and g + 64, and of the tile's last row
+      constexpr int RPT = kPairs / kGather;                // rows whose token this thread looks up
+      auto tile_pids = [&](int t, int (&a)[RPT], int& last) {       // ids of rows g, g + kGather, ..., and of the tile's last row
         const int t0 = g0 + t * kPairs, nq = min(kPairs, g1 - t0);
-        a = (t < ntiles && g < nq) ? __ldg(pr + t0 + g) : -1;
-        b = (t < ntiles && g + kGather < nq) ? __ldg(pr + t0 + g + kGather) : -1;
+#pragma unroll
+        for (int u = 0; u < RPT; ++u) a[u] = (t < ntiles && g + u * kGather < nq) ? __ldg(pr + t0 + g + u * kGather) : -1;
         last = t < ntiles ? __ldg(pr + t0 + nq - 1) : 0;
       };
-      int pa, pb, last;
-      tile_pids(tile, pa, pb, last);
+      int pa[RPT], last;
+      tile_pids(tile, pa, last);
       for (; tile < ntiles; tile += nsub) {
-        int pa_n, pb_n, last_n;
-        tile_pids(tile + nsub, pa_n, pb_n, last_n);
+        int pa_n[RPT], last_n;
+        tile_pids(tile + nsub, pa_n, last_n);
         const int nk = visible(last, kc);
         if (nk > 0) {
           if (nproc > 0) wait(&bars.q_empty, (nproc - 1) & 1);   // the previous tile's first product has read the buffer
-          tok_s[g] = pa >= 0 ? pa / dm.m : -1;
-          tok_s[g + kGather] = pb >= 0 ? pb / dm.m : -1;
+#pragma unroll
+          for (int u = 0; u < RPT; ++u) tok_s[g + u * kGather] = pa[u] >= 0 ? pa[u] / dm.m : -1;
           tc::named_bar_sync(1, kGather);
 #pragma unroll 4
           for (int r = g / CPR; r < kPairs; r += RPP) {
@@ -345,7 +340,9 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
           tc::named_bar_sync(1, kGather);                    // tok_s may be rewritten
           ++nproc;
         }
-        pa = pa_n; pb = pb_n; last = last_n;
+#pragma unroll
+        for (int u = 0; u < RPT; ++u) pa[u] = pa_n[u];
+        last = last_n;
       }
     }
   }
