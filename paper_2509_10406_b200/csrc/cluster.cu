@@ -320,53 +320,88 @@ k_assign(const T* __restrict__ X, int N, int C, const float* __restrict__ centre
   }
 }
 
-// Centre update: mean of the members, summed in bucket order with a fixed reduction tree, so
-// the result does not depend on scheduling.  An empty cluster keeps its centre.
+// Centre update: mean of the members, summed with a fixed reduction tree (slot s of the CTA adds members
+// s, s + SLOTS, ... in bucket order, then the slots are added in order), so the result does not depend
+// on scheduling.  An empty cluster keeps its centre.  One 256-thread CTA per cluster; a lane owns 16 bytes
+// of a row, and every slot keeps four row loads in flight (the member list is an indirection, so a
+// single load per slot leaves the kernel waiting on memory latency).
+constexpr int kUpdThreads = 256;
+
+__device__ __forceinline__ void ld16f(const float* p, float (&x)[4]) { const float4 v = *reinterpret_cast<const float4*>(p); x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w; }
+__device__ __forceinline__ void ld16f(const __nv_bfloat16* p, float (&x)[8]) {
+  const uint4 u = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int k = 0; k < 4; ++k) { x[2 * k] = __uint_as_float(w[k] << 16); x[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u); }
+}
+
 template <class T, int D>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(kUpdThreads)
 k_update(const T* __restrict__ X, int N, int C, int S, int kind, const int32_t* __restrict__ off,
          const int32_t* __restrict__ perm, float* __restrict__ centres, float* __restrict__ cnorm) {
-  constexpr int LPR = D / 4;            // lanes per row
-  constexpr int RPW = 32 / LPR;         // rows per warp step
-  constexpr int SLOTS = 4 * RPW;
-  __shared__ float4 part[SLOTS][LPR];
+  constexpr int VEC = 16 / (int)sizeof(T);     // elements per lane
+  constexpr int LPR = D / VEC;                 // lanes per row
+  constexpr int RPW = 32 / LPR;                // rows per warp step
+  constexpr int SLOTS = (kUpdThreads / 32) * RPW;
+  __shared__ float part[SLOTS][D];
+  __shared__ float n2_s[kUpdThreads / 32];
   const int c = blockIdx.x, prob = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int sub = lane / LPR, q = lane % LPR;
   const int slot = warp * RPW + sub;
-  const T* Xp = X + (size_t)prob * N * D;
+  const T* Xp = X + (size_t)prob * N * D + q * VEC;
   const int32_t* o = off + (size_t)prob * (C * S + 1);
   const int32_t* pm = perm + (size_t)prob * N;
-  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  float s[VEC];
+#pragma unroll
+  for (int k = 0; k < VEC; ++k) s[k] = 0.f;
   int count = 0;
   const int nranges = kind == 0 ? S : 1;
   for (int r = 0; r < nranges; ++r) {
-    int p0 = kind == 0 ? o[r * C + c] : o[c * S];
-    int p1 = kind == 0 ? o[r * C + c + 1] : o[(c + 1) * S];
+    const int p0 = kind == 0 ? o[r * C + c] : o[c * S];
+    const int p1 = kind == 0 ? o[r * C + c + 1] : o[(c + 1) * S];
     count += p1 - p0;
-    for (int p = p0 + slot; p < p1; p += SLOTS) {
-      float4 v = ld4(Xp + (size_t)pm[p] * D + q * 4);
-      s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    for (int p = p0 + slot; p < p1; p += 4 * SLOTS) {
+      int idx[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) idx[u] = p + u * SLOTS < p1 ? pm[p + u * SLOTS] : -1;
+      float v[4][VEC];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (idx[u] >= 0) ld16f(Xp + (size_t)idx[u] * D, v[u]);
+        else {
+#pragma unroll
+          for (int k = 0; k < VEC; ++k) v[u][k] = 0.f;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+#pragma unroll
+        for (int k = 0; k < VEC; ++k) s[k] += v[u][k];
     }
   }
-  part[slot][q] = s;
+#pragma unroll
+  for (int k = 0; k < VEC; ++k) part[slot][q * VEC + k] = s[k];
   __syncthreads();
-  if (threadIdx.x < 32) {
-    float4 tot = make_float4(0.f, 0.f, 0.f, 0.f);
-    float* dst = centres + ((size_t)prob * C + c) * D;
-    if (lane < LPR) {
-      for (int k = 0; k < SLOTS; ++k) { float4 v = part[k][lane]; tot.x += v.x; tot.y += v.y; tot.z += v.z; tot.w += v.w; }
-      if (count > 0) {
-        float inv = 1.f / (float)count;
-        tot.x *= inv; tot.y *= inv; tot.z *= inv; tot.w *= inv;
-        st4(dst + lane * 4, tot);
-      } else {
-        tot = ld4(dst + lane * 4);
-      }
-    }
-    float n2 = tot.x * tot.x + tot.y * tot.y + tot.z * tot.z + tot.w * tot.w;
-    n2 = warp_sum(n2);
-    if (lane == 0) cnorm[(size_t)prob * C + c] = n2;
+  float n2 = 0.f;
+  if (threadIdx.x < D) {
+    const int d = threadIdx.x;
+    float tot = 0.f;
+    float* dst = centres + ((size_t)prob * C + c) * D + d;
+#pragma unroll
+    for (int k = 0; k < SLOTS; ++k) tot += part[k][d];
+    if (count > 0) { tot *= 1.f / (float)count; *dst = tot; }
+    else tot = *dst;
+    n2 = tot * tot;
+  }
+  n2 = warp_sum(n2);
+  if (lane == 0) n2_s[warp] = n2;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+#pragma unroll
+    for (int k = 0; k < D / 32; ++k) t += n2_s[k];
+    cnorm[(size_t)prob * C + c] = t;
   }
 }
 
@@ -407,7 +442,7 @@ static int lloyd_t(const Dims& d, const T* X, int problems, int C, int kind, con
     int rc = bucket_sort(0, assign, problems, d.N, C, d.S, d.Bs, kind, off, perm, scratch, st);
     if (rc != MUSE_OK) return rc;
     prof_mark("k_update", st);
-    k_update<T, D><<<dim3(C, problems), 128, 0, st>>>(X, d.N, C, d.S, kind, off, perm, centres, cnorm);
+    k_update<T, D><<<dim3(C, problems), kUpdThreads, 0, st>>>(X, d.N, C, d.S, kind, off, perm, centres, cnorm);
     MUSE_LAUNCH_OK();
   }
   return MUSE_OK;

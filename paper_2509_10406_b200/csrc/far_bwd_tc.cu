@@ -1,4 +1,4 @@
-// Far-field backward on the tensor cores (bf16 mode, D = 128, Ck a multiple of 128, <= 2048).
+// Far-field backward on the tensor cores (bf16 mode, D = 64 or 128, Ck a multiple of 128, <= 2048).
 // One CTA per (query cluster i, plane, head) segment.  Clusters sit on the MMA M side (128 per
 // tile, one TMEM lane each), the segment's queries on the N side (64 per sweep; a longer segment
 // takes further sweeps that add to the stored gradients).  Per cluster tile, with L the merged log-sum-exp and delta = dO.O:
@@ -21,17 +21,19 @@ int make_tmap_bf16_nd(void* out_map, const void* base, int rank, const uint64_t*
                       const uint32_t* box);
 
 namespace fb {
-constexpr int D = 128, TJ = 128, NR = 64, NP = 1;
+constexpr int TJ = 128, NR = 64, NP = 1;
 constexpr int THREADS = 288, CW = 256, ISSUER = 256;   // warps 0-7 do the arithmetic; lane 0 of a ninth warp issues every TMA transfer and MMA
-constexpr int kTile = TJ * D * 2;                 // 32 KB operand tile [128][128] bf16
-constexpr int kRows = NR * D * 2;                 // 16 KB tile of 64 query rows
-constexpr int oHi = 0, oLo = oHi + kTile, oNu = oLo + kTile;
-constexpr int oQ = oNu + kTile, oDO = oQ + NP * kRows;
-constexpr int oPt = oDO + NP * kRows, oGt = oPt + TJ * NR * 2;
-// gradient rows on their way out: dkappa is staged in the (consumed) P / G tiles, dnu in a tile of its own,
-// so that the three operand tiles are free for the next cluster tile as soon as the MMAs have finished
-constexpr int oStK = oPt, oStN = oGt + TJ * NR * 2;
-constexpr int oMask = oStN + kTile;               // [NP*NR rows][Ck/32] words follow
+template <int D> struct Lay {
+  static constexpr int kTile = TJ * D * 2;        // operand tile [128 clusters][D] bf16
+  static constexpr int kRows = NR * D * 2;        // tile of 64 query rows
+  static constexpr int oHi = 0, oLo = oHi + kTile, oNu = oLo + kTile;
+  static constexpr int oQ = oNu + kTile, oDO = oQ + NP * kRows;
+  static constexpr int oPt = oDO + NP * kRows, oGt = oPt + TJ * NR * 2;
+  // gradient rows on their way out: dkappa is staged in the (consumed) P / G tiles, dnu in a tile of its own,
+  // so that the three operand tiles are free for the next cluster tile as soon as the MMAs have finished
+  static constexpr int oStK = oPt, oStN = oGt + TJ * NR * 2;
+  static constexpr int oMask = oStN + kTile;      // [NP*NR rows][Ck/32] words follow
+};
 constexpr uint32_t cS = 0, cDP = 64, cDNU = 128, cDKA = 256, cDQ = 384;   // TMEM columns
 constexpr float kLog2e = 1.4426950408889634f;
 }  // namespace fb
@@ -42,6 +44,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+template <int D>
 __global__ void __launch_bounds__(fb::THREADS, 1)
 k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_constant__ CUtensorMap tm_klo,
              const __grid_constant__ CUtensorMap tm_nu, const __grid_constant__ CUtensorMap tm_gka,
@@ -51,6 +54,9 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
              const float* __restrict__ beta, const float* __restrict__ mu, float* __restrict__ dQacc, bf16* __restrict__ dkappa,
              bf16* __restrict__ dnu, float* __restrict__ dS, int grad_by_key_cluster, int* __restrict__ status) {
   using namespace fb;
+  typedef Lay<D> LY;
+  constexpr int kTile = LY::kTile, kRows = LY::kRows, oHi = LY::oHi, oLo = LY::oLo, oNu = LY::oNu, oQ = LY::oQ, oDO = LY::oDO,
+                oPt = LY::oPt, oGt = LY::oGt, oStK = LY::oStK, oStN = LY::oStN, oMask = LY::oMask, G = D / 64, CPR = D / 8;
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   // bar_full: kappa tiles landed; bar_nu: nu tile landed; bar1: S / dPnu products done; bar2: dnu / dkappa
   // products done; bar3: dq products done as well; bar_st: the previous tile's stores have read their staging
@@ -72,8 +78,8 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     // [plane][j][i] layout) takes whole tiles of rows without looking at which segments exist.
     if (grad_by_key_cluster) {
       const size_t row0 = ((size_t)pq * dm.SB + pl) * Ck;
-      for (int e = tid; e < Ck * (D / 8); e += blockDim.x) {
-        const size_t at = ((row0 + (e >> 4)) * dm.Cq + i) * D + (e & 15) * 8;
+      for (int e = tid; e < Ck * CPR; e += blockDim.x) {
+        const size_t at = ((row0 + (e / CPR)) * dm.Cq + i) * D + (e % CPR) * 8;
         *reinterpret_cast<uint4*>(dkappa + at) = make_uint4(0u, 0u, 0u, 0u);
         *reinterpret_cast<uint4*>(dnu + at) = make_uint4(0u, 0u, 0u, 0u);
       }
@@ -105,13 +111,15 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   auto issue_kappa = [&](int jt_) {                       // issuer: the two kappa tiles of cluster tile jt_
     tc::mbar_expect_tx(&bar_full, 2 * kTile);
     const int row = (int)(ent0 + (size_t)jt_ * TJ);
-    tc::tma_load_2d(sm + oHi, &tm_khi, 0, row, &bar_full); tc::tma_load_2d(sm + oHi + TJ * 128, &tm_khi, 64, row, &bar_full);
-    tc::tma_load_2d(sm + oLo, &tm_klo, 0, row, &bar_full); tc::tma_load_2d(sm + oLo + TJ * 128, &tm_klo, 64, row, &bar_full);
+    for (int g = 0; g < G; ++g) {
+      tc::tma_load_2d(sm + oHi + g * TJ * 128, &tm_khi, 64 * g, row, &bar_full);
+      tc::tma_load_2d(sm + oLo + g * TJ * 128, &tm_klo, 64 * g, row, &bar_full);
+    }
   };
   auto issue_nu = [&](int jt_) {                          // issuer: its nu tile
     tc::mbar_expect_tx(&bar_nu, kTile);
     const int row = (int)(ent0 + (size_t)jt_ * TJ);
-    tc::tma_load_2d(sm + oNu, &tm_nu, 0, row, &bar_nu); tc::tma_load_2d(sm + oNu + TJ * 128, &tm_nu, 64, row, &bar_nu);
+    for (int g = 0; g < G; ++g) tc::tma_load_2d(sm + oNu + g * TJ * 128, &tm_nu, 64 * g, row, &bar_nu);
   };
   for (int s0 = p0; s0 < p1 && ok; s0 += NP * NR) {        // sweep: up to 64 rows
     const int ns = min(NP * NR, p1 - s0), np = (ns + NR - 1) / NR;
@@ -127,8 +135,8 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     }
     for (int e = tid; e < 2 * Ck; e += THREADS) smask[e] = 0u;
     __syncthreads();
-    for (int e = tid; e < NP * NR * (D / 8); e += THREADS) {
-      const int r = e >> 4, ck = e & 15, kb = ck >> 3, c = ck & 7, p = r / NR, rr = r % NR;
+    for (int e = tid; e < NP * NR * CPR; e += THREADS) {
+      const int r = e / CPR, ck = e % CPR, kb = ck >> 3, c = ck & 7, p = r / NR, rr = r % NR;
       uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
       if (r < ns) {
         a = reinterpret_cast<const uint4*>(Qp + (size_t)rows[r] * D)[ck];
@@ -263,7 +271,9 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
         if (tid == ISSUER) {
           tc::fence_after_sync();
           const uint32_t id_row = tc::idesc_bf16(TJ, D, 0, 1);      // A K-major (P / G), B = query rows, MN-major
-          const uint32_t id_dq = tc::idesc_bf16(D, NR, 1, 1);       // A = kappa tile MN-major, B = G MN-major
+          // A = kappa tile MN-major, B = G MN-major.  M = 128 output dims even when D = 64: the second 64-dim group of the
+          // operand is then the tile that follows in shared memory, and output lanes 64..127 hold numbers that nobody reads
+          const uint32_t id_dq = tc::idesc_bf16(128, NR, 1, 1);
 #pragma unroll
           for (int ks = 0; ks < NR / 16; ++ks)
             tc::mma_bf16_ss(tbase + cDNU, tc::smem_desc_sw128(aPt + ks * 32, 16, 1024),
@@ -361,11 +371,15 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
         const int c1 = grad_by_key_cluster ? i : 0;
         const int c2 = grad_by_key_cluster ? (pq * dm.SB + pl) * Ck + jt * TJ : (int)(ent0 + (size_t)jt * TJ);
         if (!later_sweep) {
-          tc::tma_store_3d(&tm_gnu, sm + oStN, 0, c1, c2); tc::tma_store_3d(&tm_gnu, sm + oStN + TJ * 128, 64, c1, c2);
-          tc::tma_store_3d(&tm_gka, sm + oStK, 0, c1, c2); tc::tma_store_3d(&tm_gka, sm + oStK + TJ * 128, 64, c1, c2);
+          for (int g = 0; g < G; ++g) {
+            tc::tma_store_3d(&tm_gnu, sm + oStN + g * TJ * 128, 64 * g, c1, c2);
+            tc::tma_store_3d(&tm_gka, sm + oStK + g * TJ * 128, 64 * g, c1, c2);
+          }
         } else {                              // a further sweep of a long segment adds to the stored rows
-          tc::tma_reduce_add_3d(&tm_gnu, sm + oStN, 0, c1, c2); tc::tma_reduce_add_3d(&tm_gnu, sm + oStN + TJ * 128, 64, c1, c2);
-          tc::tma_reduce_add_3d(&tm_gka, sm + oStK, 0, c1, c2); tc::tma_reduce_add_3d(&tm_gka, sm + oStK + TJ * 128, 64, c1, c2);
+          for (int g = 0; g < G; ++g) {
+            tc::tma_reduce_add_3d(&tm_gnu, sm + oStN + g * TJ * 128, 64 * g, c1, c2);
+            tc::tma_reduce_add_3d(&tm_gka, sm + oStK + g * TJ * 128, 64 * g, c1, c2);
+          }
         }
         tc::tma_store_commit();
       }
@@ -388,7 +402,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       for (int c0 = 32 * wg; c0 < NR; c0 += 64) {
         float v[32];
         tc::tmem_ld32(tlane + cDQ + p * NR + c0, v);
-        if (ok) {
+        if (ok && L < D) {
 #pragma unroll
           for (int r = 0; r < 32; ++r) {
             const int rr = p * NR + c0 + r;
@@ -413,7 +427,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 
 bool far_bwd_tc_supported(const Dims& d, int dtype) {
   // (the far-set mask, 8 bytes per key cluster, shares the CTA's shared memory with 200 KB of tiles)
-  return dtype == MUSE_BF16 && d.D == fb::D && d.Ck % fb::TJ == 0 && d.Ck <= 2048;
+  return dtype == MUSE_BF16 && (d.D == 64 || d.D == 128) && d.Ck % fb::TJ == 0 && d.Ck <= 2048;
 }
 
 int far_bwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const void* dO, const float* qbar, const float* LSE,
@@ -421,25 +435,35 @@ int far_bwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const void* dO,
                void* dkappa, void* dnu, float* dS, int grad_by_key_cluster, int* status, cudaStream_t st) {
   const uint64_t ent = (uint64_t)d.B * d.Hq * d.SB * d.Cq * d.Ck;
   CUtensorMap khi, klo, nu;
-  int rc = make_tmap_bf16_rows(&khi, sp.khi, ent, fb::D, fb::TJ);
-  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&klo, sp.klo, ent, fb::D, fb::TJ);
-  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&nu, sp.nu, ent, fb::D, fb::TJ);
+  const uint64_t Dd = (uint64_t)d.D;
+  int rc = make_tmap_bf16_rows(&khi, sp.khi, ent, d.D, fb::TJ);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&klo, sp.klo, ent, d.D, fb::TJ);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&nu, sp.nu, ent, d.D, fb::TJ);
   // gradient tensors for the tiled stores: (d, i, plane * Ck + j) when grouped by key cluster, else (d, 1, entry)
   CUtensorMap gka, gnu;
   const uint64_t rows_j = (uint64_t)d.B * d.Hq * d.SB * d.Ck;
-  const uint64_t dims_a[3] = {(uint64_t)fb::D, (uint64_t)d.Cq, rows_j}, str_a[2] = {(uint64_t)fb::D * 2, (uint64_t)d.Cq * fb::D * 2};
-  const uint64_t dims_b[3] = {(uint64_t)fb::D, 1, ent}, str_b[2] = {(uint64_t)fb::D * 2, (uint64_t)fb::D * 2};
+  const uint64_t dims_a[3] = {Dd, (uint64_t)d.Cq, rows_j}, str_a[2] = {Dd * 2, (uint64_t)d.Cq * Dd * 2};
+  const uint64_t dims_b[3] = {Dd, 1, ent}, str_b[2] = {Dd * 2, Dd * 2};
   const uint32_t box[3] = {64, 1, (uint32_t)fb::TJ};
   if (rc == MUSE_OK) rc = make_tmap_bf16_nd(&gka, dkappa, 3, grad_by_key_cluster ? dims_a : dims_b, grad_by_key_cluster ? str_a : str_b, box);
   if (rc == MUSE_OK) rc = make_tmap_bf16_nd(&gnu, dnu, 3, grad_by_key_cluster ? dims_a : dims_b, grad_by_key_cluster ? str_a : str_b, box);
   if (rc != MUSE_OK) return rc;
   if (ent >= (1ull << 31)) return MUSE_ERR_UNSUPPORTED;      // 32-bit tile coordinates
-  const size_t smem = (size_t)fb::oMask + (size_t)fb::NP * fb::NR * (d.Ck / 32) * 4 + 1024;
-  MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_bwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const size_t mask_bytes = (size_t)fb::NP * fb::NR * (d.Ck / 32) * 4;
   prof_mark("k_far_bwd_tc", st);
-  k_far_bwd_tc<<<dim3(d.Cq, d.SB, d.B * d.Hq), fb::THREADS, smem, st>>>(
-      d, khi, klo, nu, gka, gnu, (const bf16*)Q, (const bf16*)dO, qbar, LSE, delta, off_q, perm_q, sel, sp.beta, sp.mu, dQacc, (bf16*)dkappa,
-      (bf16*)dnu, dS, grad_by_key_cluster, status);
+  if (d.D == 128) {
+    const size_t smem = (size_t)fb::Lay<128>::oMask + mask_bytes + 1024;
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_bwd_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k_far_bwd_tc<128><<<dim3(d.Cq, d.SB, d.B * d.Hq), fb::THREADS, smem, st>>>(
+        d, khi, klo, nu, gka, gnu, (const bf16*)Q, (const bf16*)dO, qbar, LSE, delta, off_q, perm_q, sel, sp.beta, sp.mu, dQacc, (bf16*)dkappa,
+        (bf16*)dnu, dS, grad_by_key_cluster, status);
+  } else {
+    const size_t smem = (size_t)fb::Lay<64>::oMask + mask_bytes + 1024;
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_bwd_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k_far_bwd_tc<64><<<dim3(d.Cq, d.SB, d.B * d.Hq), fb::THREADS, smem, st>>>(
+        d, khi, klo, nu, gka, gnu, (const bf16*)Q, (const bf16*)dO, qbar, LSE, delta, off_q, perm_q, sel, sp.beta, sp.mu, dQacc, (bf16*)dkappa,
+        (bf16*)dnu, dS, grad_by_key_cluster, status);
+  }
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }

@@ -1,4 +1,4 @@
-// Far-field forward on the tensor cores (bf16 mode, D = 128, Ck a multiple of 128, Ck <= 2048).
+// Far-field forward on the tensor cores (bf16 mode, D = 64 or 128, Ck a multiple of 128, Ck <= 2048).
 // One CTA per (query cluster i, plane, head) segment; its queries (32 on average at the headline
 // sizes, up to 64 per pass) share the Ck accumulated summaries of (i, plane).  The summaries sit
 // on the MMA M side (128 clusters per tile, one TMEM lane each) and the queries on the N side
@@ -20,11 +20,10 @@ namespace muse {
 typedef __nv_bfloat16 bf16;
 int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
 
-constexpr int kFD = 128, kFJ = 128;                 // head dim, clusters per tile
+constexpr int kFJ = 128;                            // clusters per tile
 // Queries per pass FR and per selection step FQ (one warp each) are template parameters: 64 / 16 up to 1024
 // key clusters, 32 / 8 up to 2048 (all FR x Ck scores of a pass live in the 512 TMEM columns, P and the score
 // rows of a step in shared memory).
-constexpr int kTileBytes = kFJ * kFD * 2;           // 32 KB: one [128][128] bf16 operand tile
 constexpr int kFarTcCols = 512;
 constexpr int kMaxStA = 6, kMaxStD = 4;
 constexpr int kCandMax = 128;                       // candidates kept by the compacting selection (4 per lane)
@@ -222,7 +221,7 @@ __device__ __forceinline__ void select_top_m(float* s, int Ck, int m, int32_t* s
   for (int k = base + lane; k < m; k += 32) so[k] = -1;
 }
 
-template <int FR, int FQ>
+template <int FR, int FQ, int D>
 __global__ void __launch_bounds__(FQ * 32, 1)
 k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_constant__ CUtensorMap tm_klo,
              const __grid_constant__ CUtensorMap tm_nu, const bf16* __restrict__ Q, const int32_t* __restrict__ off_q,
@@ -230,6 +229,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
              const int32_t* __restrict__ sel_in, int32_t* __restrict__ sel_out, float* __restrict__ o_far,
              float* __restrict__ lse_far, int p_bytes, int sc_bytes, int nsA, int nsD, int* __restrict__ status) {
   constexpr int NT = FQ * 32, NTG = FQ / 4, KT = 16 / NTG;   // threads; tile groups in the TMEM read-out; cluster tiles per group
+  constexpr int kTileBytes = kFJ * D * 2, G = D / 64;        // one [128 clusters][D] bf16 operand tile; 128-byte column groups of a row
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ FarBars bars;
   __shared__ uint32_t tbase_s;
@@ -251,7 +251,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   const size_t ent0 = (((size_t)pq * dm.SB + pl) * dm.Cq + i) * Ck;
   const float* mup = mu + ent0;
   const float* bep = beta + ent0;
-  const bf16* Qp = Q + (size_t)pq * dm.N * kFD;
+  const bf16* Qp = Q + (size_t)pq * dm.N * D;
   const int32_t* pm = perm_q + (size_t)pq * dm.N;
 
   if (warp == 0) tc::tmem_alloc(&tbase_s, kFarTcCols);
@@ -316,19 +316,18 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       tc::mbar_expect_tx(&bars.fullA[s], kTileBytes);
       const void* map = (t & 1) ? (const void*)&tm_klo : (const void*)&tm_khi;
       const int row = (int)(ent0 + (size_t)(t >> 1) * kFJ);
-      tc::tma_load_2d(sm + s * kTileBytes, map, 0, row, &bars.fullA[s]);
-      tc::tma_load_2d(sm + s * kTileBytes + kFJ * 128, map, 64, row, &bars.fullA[s]);
+      for (int g = 0; g < G; ++g) tc::tma_load_2d(sm + s * kTileBytes + g * kFJ * 128, map, 64 * g, row, &bars.fullA[s]);
     };
     const int TA = 2 * NJ, TA0 = min(nsA, TA);
     if (prod >= 0 && prod < WA)
       for (int t = 0; t < TA0 && ok; ++t, next_a())
         if (wa == prod) produce_a(t);
     if (tid < FR) rows[tid] = tid < n ? pm[r0 + tid] : -1;
-    // query rows -> K-major swizzled tile [64][128] bf16 (2 blocks of [64][128 B])
-    for (int e = tid; e < FR * (kFD / 8); e += NT) {
-      const int r = e >> 4, ck = e & 15, kb = ck >> 3, c = ck & 7;
+    // query rows -> K-major swizzled tile [FR][D] bf16 (G blocks of [FR][128 B])
+    for (int e = tid; e < FR * (D / 8); e += NT) {
+      const int r = e / (D / 8), ck = e % (D / 8), kb = ck >> 3, c = ck & 7;
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (r < n) v = reinterpret_cast<const uint4*>(Qp + (size_t)pm[r0 + r] * kFD)[ck];
+      if (r < n) v = reinterpret_cast<const uint4*>(Qp + (size_t)pm[r0 + r] * D)[ck];
       *reinterpret_cast<uint4*>(Qs + kb * FR * 128 + tc::sw128_off(r, c)) = v;
     }
     tc::fence_async_smem();
@@ -340,8 +339,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
           if (wa == prod) produce_a(t);
       // bring the nu tiles of this segment into L2 while the selection runs
       for (int t = prod; t < NJ; t += 4) {
-        tc::tma_prefetch_2d(&tm_nu, 0, (int)(ent0 + (size_t)t * kFJ));
-        tc::tma_prefetch_2d(&tm_nu, 64, (int)(ent0 + (size_t)t * kFJ));
+        for (int g = 0; g < G; ++g) tc::tma_prefetch_2d(&tm_nu, 64 * g, (int)(ent0 + (size_t)t * kFJ));
       }
     } else if (tid == 32) {
       tc::fence_after_sync();
@@ -363,7 +361,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
         const uint32_t dcol = tbase + (u >> 1) * FR;
 
 #pragma unroll
-        for (int ks = 0; ks < kFD / 16; ++ks)
+        for (int ks = 0; ks < D / 16; ++ks)
           tc::mma_bf16_ss(dcol, tc::desc_step(da, (ks / 4) * kFJ * 128 + (ks % 4) * 32),
                           tc::desc_step(dq0, (ks / 4) * FR * 128 + (ks % 4) * 32), idesc, (u & 1) || ks > 0);
         tc::mma_commit(&bars.emptyA[s]);
@@ -479,12 +477,13 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
         if (!tc::mbar_wait(&bars.emptyD[s_], ph_ ^ 1)) { ok = false; break; }
         tc::mbar_expect_tx(&bars.fullD[s_], kTileBytes);
         const int row = (int)(ent0 + (size_t)t * kFJ);
-        tc::tma_load_2d(ring + s_ * kTileBytes, &tm_nu, 0, row, &bars.fullD[s_]);
-        tc::tma_load_2d(ring + s_ * kTileBytes + kFJ * 128, &tm_nu, 64, row, &bars.fullD[s_]);
+        for (int g = 0; g < G; ++g) tc::tma_load_2d(ring + s_ * kTileBytes + g * kFJ * 128, &tm_nu, 64 * g, row, &bars.fullD[s_]);
       }
     } else if (tid == 32 && ok) {
       tc::fence_after_sync();
-      const uint32_t idesc = tc::idesc_bf16(kFD, FR, 1, 0);
+      // M = 128 output dims even when D = 64: the second 64-dim group of the MN-major operand then reads whatever
+      // follows the tile in shared memory, and output lanes 64..127 hold numbers that nobody reads
+      const uint32_t idesc = tc::idesc_bf16(128, FR, 1, 0);
       const uint64_t dp0 = tc::smem_desc_sw128(tc::smem_u32(Pm), 16, 1024);
       const uint64_t dn0 = tc::smem_desc_sw128(tc::smem_u32(sm + p_bytes), kFJ * 128, 1024);
 #ifdef MUSE_PHASE_CLOCKS
@@ -528,10 +527,10 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
       const int half = warp >> 2;
       float v[32];
       tc::tmem_ld32(tbase + ((uint32_t)(lq * 32) << 16) + 32 * half, v);
-      if (ok) {
+      if (ok && (tid & 127) < D) {
 #pragma unroll
         for (int r = 0; r < 32; ++r)
-          if (32 * half + r < n) o_far[((size_t)pq * dm.N + rows[32 * half + r]) * kFD + (tid & 127)] = v[r] * rinv[32 * half + r];
+          if (32 * half + r < n) o_far[((size_t)pq * dm.N + rows[32 * half + r]) * D + (tid & 127)] = v[r] * rinv[32 * half + r];
       }
     }
     tc::fence_before_sync();
@@ -544,36 +543,38 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 }
 
 bool far_fwd_tc_supported(const Dims& d, int dtype) {
-  return dtype == MUSE_BF16 && d.D == kFD && d.Ck % kFJ == 0 && d.Ck <= 2048 && d.Ck >= kFJ;
+  return dtype == MUSE_BF16 && (d.D == 64 || d.D == 128) && d.Ck % kFJ == 0 && d.Ck <= 2048 && d.Ck >= kFJ;
 }
 
 int far_fwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const int32_t* off_q, const int32_t* perm_q,
                const int32_t* sel_in, int32_t* sel_out, float* o_far, float* lse_far, int* status, cudaStream_t st) {
   const uint64_t ent = (uint64_t)d.B * d.Hq * d.SB * d.Cq * d.Ck;
   CUtensorMap khi, klo, nu;
-  int rc = make_tmap_bf16_rows(&khi, sp.khi, ent, kFD, kFJ);
-  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&klo, sp.klo, ent, kFD, kFJ);
-  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&nu, sp.nu, ent, kFD, kFJ);
+  int rc = make_tmap_bf16_rows(&khi, sp.khi, ent, d.D, kFJ);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&klo, sp.klo, ent, d.D, kFJ);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&nu, sp.nu, ent, d.D, kFJ);
   if (rc != MUSE_OK) return rc;
   const bool wide = d.Ck > 1024;                                         // 32 queries per pass, 8 per selection step
   const int FR = wide ? 32 : 64, FQ = wide ? 8 : 16;
+  const int tile_bytes = kFJ * d.D * 2;
   const int p_bytes = FR * d.Ck * 2;                                     // P: bf16 [FR][Ck]
   int sc_bytes = FQ * d.Ck * 4;                                          // FQ score rows, later the nu ring
-  if (sc_bytes < 2 * kTileBytes) sc_bytes = 2 * kTileBytes;
-  int nsA = (p_bytes + sc_bytes) / kTileBytes, nsD = sc_bytes / kTileBytes;
+  if (sc_bytes < 2 * tile_bytes) sc_bytes = 2 * tile_bytes;
+  int nsA = (p_bytes + sc_bytes) / tile_bytes, nsD = sc_bytes / tile_bytes;
   nsA = nsA > kMaxStA ? kMaxStA : nsA;
   nsD = nsD > kMaxStD ? kMaxStD : nsD;
-  const size_t smem = (size_t)p_bytes + sc_bytes + FR * kFD * 2 + 1024;
+  // (D = 64: one more tile of room behind the ring, which the padded 128-row products of phase D read past)
+  const size_t smem = (size_t)p_bytes + sc_bytes + FR * d.D * 2 + 1024 + (d.D == 64 ? tile_bytes : 0);
   prof_mark("k_far_fwd_tc", st);
-  if (wide) {
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_fwd_tc<32, 8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_far_fwd_tc<32, 8><<<dim3(d.Cq, d.SB, d.B * d.Hq), 256, smem, st>>>(d, khi, klo, nu, (const bf16*)Q, off_q, perm_q, sp.mu, sp.beta,
-                                                                 sel_in, sel_out, o_far, lse_far, p_bytes, sc_bytes, nsA, nsD, status);
-  } else {
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_fwd_tc<64, 16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_far_fwd_tc<64, 16><<<dim3(d.Cq, d.SB, d.B * d.Hq), 512, smem, st>>>(d, khi, klo, nu, (const bf16*)Q, off_q, perm_q, sp.mu, sp.beta,
-                                                                   sel_in, sel_out, o_far, lse_far, p_bytes, sc_bytes, nsA, nsD, status);
-  }
+#define MUSE_FAR_FWD_LAUNCH(FR_, FQ_, D_)                                                                                   \
+  do {                                                                                                                    \
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_fwd_tc<FR_, FQ_, D_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+    k_far_fwd_tc<FR_, FQ_, D_><<<dim3(d.Cq, d.SB, d.B * d.Hq), FQ_ * 32, smem, st>>>(                                       \
+        d, khi, klo, nu, (const bf16*)Q, off_q, perm_q, sp.mu, sp.beta, sel_in, sel_out, o_far, lse_far, p_bytes, sc_bytes, nsA, nsD, status); \
+  } while (0)
+  if (wide) { if (d.D == 128) MUSE_FAR_FWD_LAUNCH(32, 8, 128); else MUSE_FAR_FWD_LAUNCH(32, 8, 64); }
+  else { if (d.D == 128) MUSE_FAR_FWD_LAUNCH(64, 16, 128); else MUSE_FAR_FWD_LAUNCH(64, 16, 64); }
+#undef MUSE_FAR_FWD_LAUNCH
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }

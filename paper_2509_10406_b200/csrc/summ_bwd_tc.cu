@@ -1,5 +1,5 @@
 // Key-side pass of the backward through the accumulated summaries, on the tensor cores
-// (bf16 mode, D = 128, Cq a multiple of 128).  One CTA per (key cluster j, head).  For every
+// (bf16 mode, D = 64 or 128, Cq a multiple of 8).  One CTA per (key cluster j, head).  For every
 // plane pl the summary (i, j, pl) was built from the keys u of cluster j in blocks <= pl, with
 // weights w_iu = exp(sigma qbar_i.k_u - mu_ij(pl)) <= 1.  Given the far-field gradients
 // (dkappa, dnu, dS) of that plane:
@@ -20,21 +20,24 @@ namespace muse {
 typedef __nv_bfloat16 bf16;
 
 namespace sb {
-constexpr int D = 128, TI = 128, NU = 64;
+constexpr int TI = 128, NU = 64;
 constexpr int THREADS = 288, ISSUER = 256;     // warps 0-7 do the arithmetic; lane 0 of a ninth warp issues every TMA load and MMA
-constexpr int kTile = TI * D * 2;              // 32 KB
-constexpr int kKeys = NU * D * 2;              // 16 KB
-// The low half of the centroid tile is only needed for the tilt logits, which do not depend on
-// the plane: once they are in TMEM its space serves as the second dkappa buffer.
-constexpr int oQhi = 0, oQlo = oQhi + kTile, oDka0 = oQlo + kTile, oDnu0 = oDka0 + kTile, oDnu1 = oDnu0 + kTile;
-constexpr int oK = oDnu1 + kTile, oV = oK + kKeys, oW = oV + kKeys, oWc = oW + TI * NU * 2;
-constexpr int total = oWc + TI * NU * 2 + 1024;
+template <int D> struct Lay {
+  static constexpr int kTile = TI * D * 2;     // [128 query clusters][D] bf16
+  static constexpr int kKeys = NU * D * 2;     // [64 keys][D] bf16
+  // The low half of the centroid tile is only needed for the tilt logits, which do not depend on
+  // the plane: once they are in TMEM its space serves as the second dkappa buffer.
+  static constexpr int oQhi = 0, oQlo = oQhi + kTile, oDka0 = oQlo + kTile, oDnu0 = oDka0 + kTile, oDnu1 = oDnu0 + kTile;
+  static constexpr int oK = oDnu1 + kTile, oV = oK + kKeys, oW = oV + kKeys, oWc = oW + TI * NU * 2;
+  static constexpr int total = oWc + TI * NU * 2 + 1024;
+};
 constexpr uint32_t cL = 0, cX1 = 64, cX2 = 128, cDK = 192, cDV = 256;
 }  // namespace sb
 
 // 2-D tensor map over a bf16 matrix with an arbitrary row pitch (bytes), 128B swizzle, box [box_rows][64]
 int make_tmap_bf16_pitched(void* out_map, const void* base, uint64_t rows, uint64_t cols, uint64_t pitch_bytes, uint32_t box_rows);
 
+template <int D>
 __global__ void __launch_bounds__(sb::THREADS, 1)
 k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_constant__ CUtensorMap tm_dnu,
               const __grid_constant__ CUtensorMap tm_K, const __grid_constant__ CUtensorMap tm_V,
@@ -43,6 +46,9 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
               const float* __restrict__ mu, const float* __restrict__ dS, float* __restrict__ dK_perm,
               float* __restrict__ dV_perm, int* __restrict__ status) {
   using namespace sb;
+  typedef Lay<D> LY;
+  constexpr int kTile = LY::kTile, kKeys = LY::kKeys, oQhi = LY::oQhi, oQlo = LY::oQlo, oDka0 = LY::oDka0, oDnu0 = LY::oDnu0,
+                oDnu1 = LY::oDnu1, oK = LY::oK, oV = LY::oV, oW = LY::oW, oWc = LY::oWc, G = D / 64;
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar_g[2], bar_kv, bar_q, bar_l, bar1, bar2;
   __shared__ uint32_t tbase_s;
@@ -82,8 +88,10 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
     if (tid == ISSUER) {
       tc::mbar_expect_tx(&bar_kv, 2 * kKeys);
       const int row = (int)((size_t)pk * dm.N + c0);
-      tc::tma_load_2d(sm + oK, &tm_K, 0, row, &bar_kv); tc::tma_load_2d(sm + oK + NU * 128, &tm_K, 64, row, &bar_kv);
-      tc::tma_load_2d(sm + oV, &tm_V, 0, row, &bar_kv); tc::tma_load_2d(sm + oV + NU * 128, &tm_V, 64, row, &bar_kv);
+      for (int g = 0; g < G; ++g) {
+        tc::tma_load_2d(sm + oK + g * NU * 128, &tm_K, 64 * g, row, &bar_kv);
+        tc::tma_load_2d(sm + oV + g * NU * 128, &tm_V, 64 * g, row, &bar_kv);
+      }
     }
     int pl0 = 0;                                          // planes [pl0, SB) see this chunk (bucket ends grow with the plane)
     while (pl0 < dm.SB && ok_[pl0 + 1] <= c0) ++pl0;
@@ -99,8 +107,10 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         const int row = (int)((((size_t)pq * dm.SB + pl) * dm.Ck + j) * dm.Cq + i0);
         unsigned char* dka = sm + (buf ? oQlo : oDka0);
         unsigned char* dnu = sm + (buf ? oDnu1 : oDnu0);
-        tc::tma_load_2d(dka, &tm_dka, 0, row, &bar_g[buf]); tc::tma_load_2d(dka + TI * 128, &tm_dka, 64, row, &bar_g[buf]);
-        tc::tma_load_2d(dnu, &tm_dnu, 0, row, &bar_g[buf]); tc::tma_load_2d(dnu + TI * 128, &tm_dnu, 64, row, &bar_g[buf]);
+        for (int g = 0; g < G; ++g) {
+          tc::tma_load_2d(dka + g * TI * 128, &tm_dka, 64 * g, row, &bar_g[buf]);
+          tc::tma_load_2d(dnu + g * TI * 128, &tm_dnu, 64 * g, row, &bar_g[buf]);
+        }
       };
       PCLK(7)
       __syncthreads();                                    // every MMA that read the centroid tiles has completed (bar2 waited)
@@ -108,8 +118,10 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         // sigma * qbar tile as bf16 hi + lo operands (split once per layer), and the first gradient tiles
         tc::mbar_expect_tx(&bar_q, 2 * kTile);
         const int r = pq * dm.Cq + i0;
-        tc::tma_load_2d(sm + oQhi, &tm_qhi, 0, r, &bar_q); tc::tma_load_2d(sm + oQhi + TI * 128, &tm_qhi, 64, r, &bar_q);
-        tc::tma_load_2d(sm + oQlo, &tm_qlo, 0, r, &bar_q); tc::tma_load_2d(sm + oQlo + TI * 128, &tm_qlo, 64, r, &bar_q);
+        for (int g = 0; g < G; ++g) {
+          tc::tma_load_2d(sm + oQhi + g * TI * 128, &tm_qhi, 64 * g, r, &bar_q);
+          tc::tma_load_2d(sm + oQlo + g * TI * 128, &tm_qlo, 64 * g, r, &bar_q);
+        }
         if (pl0 < dm.SB) issue_grad(pl0, 0);
       }
       // which planes hold a non-empty segment of query cluster i (others were never written by the far-field pass)
@@ -210,7 +222,9 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         __syncthreads();
         if (tid == ISSUER) {
           tc::fence_after_sync();
-          const uint32_t idesc = tc::idesc_bf16(D, NU, 1, 1);       // A [i][d] and B [i][u]: both contract over rows
+          // A [i][d] and B [i][u]: both contract over rows.  M = 128 output dims even when D = 64: the second 64-dim group
+          // of the A operand is then the tile that follows in shared memory, and output lanes 64..127 hold numbers that nobody reads
+          const uint32_t idesc = tc::idesc_bf16(128, NU, 1, 1);
 #pragma unroll
           for (int ks = 0; ks < TI / 16; ++ks)
             tc::mma_bf16_ss(tbase + cDK, tc::smem_desc_sw128(aDka + ks * 16 * 128, TI * 128, 1024),
@@ -247,7 +261,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
       float a[32], b[32];
       tc::tmem_ld32(tlane + cDK + 32 * wg, a);
       tc::tmem_ld32(tlane + cDV + 32 * wg, b);
-      if (ok && started) {
+      if (ok && started && L < D) {
 #pragma unroll
         for (int u = 0; u < 32; ++u) {
           if (32 * wg + u < nkc) {
@@ -270,7 +284,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
 }
 
 bool summ_bwd_tc_supported(const Dims& d, int dtype) {
-  return dtype == MUSE_BF16 && d.D == sb::D && d.Cq % 8 == 0;
+  return dtype == MUSE_BF16 && (d.D == 64 || d.D == 128) && d.Cq % 8 == 0;
 }
 
 int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
@@ -280,24 +294,30 @@ int summ_bwd_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* of
                 void* qsplit, int* status, cudaStream_t st) {
   // qsplit: 2 * B*Hq*Cq*D bf16 of scratch for the split centroids
   bf16* qhi = (bf16*)qsplit;
-  bf16* qlo = qhi + (size_t)d.B * d.Hq * d.Cq * sb::D;
+  bf16* qlo = qhi + (size_t)d.B * d.Hq * d.Cq * d.D;
   int rcq = split_qbar(d, qbar, qhi, qlo, st);
   if (rcq != MUSE_OK) return rcq;
   CUtensorMap tqh, tql;
-  rcq = make_tmap_bf16_rows(&tqh, qhi, (uint64_t)d.B * d.Hq * d.Cq, sb::D, sb::TI);
-  if (rcq == MUSE_OK) rcq = make_tmap_bf16_rows(&tql, qlo, (uint64_t)d.B * d.Hq * d.Cq, sb::D, sb::TI);
+  rcq = make_tmap_bf16_rows(&tqh, qhi, (uint64_t)d.B * d.Hq * d.Cq, d.D, sb::TI);
+  if (rcq == MUSE_OK) rcq = make_tmap_bf16_rows(&tql, qlo, (uint64_t)d.B * d.Hq * d.Cq, d.D, sb::TI);
   if (rcq != MUSE_OK) return rcq;
   CUtensorMap tdka, tdnu, tK, tV;
   const uint64_t grows = (uint64_t)d.B * d.Hq * d.SB * d.Ck * d.Cq;       // gradient entries, [plane][j][i]
-  int rc = make_tmap_bf16_rows(&tdka, dkappa, grows, sb::D, sb::TI);
-  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tdnu, dnu, grows, sb::D, sb::TI);
-  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tK, Kp, (uint64_t)d.B * d.Hkv * d.N, sb::D, sb::NU);
-  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tV, Vp, (uint64_t)d.B * d.Hkv * d.N, sb::D, sb::NU);
+  int rc = make_tmap_bf16_rows(&tdka, dkappa, grows, d.D, sb::TI);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tdnu, dnu, grows, d.D, sb::TI);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tK, Kp, (uint64_t)d.B * d.Hkv * d.N, d.D, sb::NU);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tV, Vp, (uint64_t)d.B * d.Hkv * d.N, d.D, sb::NU);
   if (rc != MUSE_OK) return rc;
-  MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, sb::total));
   prof_mark("k_summ_bwd_tc", st);
-  k_summ_bwd_tc<<<dim3(d.Ck, d.B * d.Hq), sb::THREADS, sb::total, st>>>(d, tdka, tdnu, tK, tV, tqh, tql, off_k, off_q, mu, dS, dK_perm,
-                                                                dV_perm, status);
+  if (d.D == 128) {
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb::Lay<128>::total));
+    k_summ_bwd_tc<128><<<dim3(d.Ck, d.B * d.Hq), sb::THREADS, sb::Lay<128>::total, st>>>(d, tdka, tdnu, tK, tV, tqh, tql, off_k, off_q, mu, dS,
+                                                                                    dK_perm, dV_perm, status);
+  } else {
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb::Lay<64>::total));
+    k_summ_bwd_tc<64><<<dim3(d.Ck, d.B * d.Hq), sb::THREADS, sb::Lay<64>::total, st>>>(d, tdka, tdnu, tK, tV, tqh, tql, off_k, off_q, mu, dS,
+                                                                                  dK_perm, dV_perm, status);
+  }
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }

@@ -22,12 +22,15 @@ int make_tmap_bf16_nd(void* out_map, const void* base, int rank, const uint64_t*
                       const uint32_t* box);
 
 namespace st {
-constexpr int D = 128, TI = 128, NU = 64, THREADS = 256;
-constexpr int kTile = TI * D * 2, kKeys = NU * D * 2, kW = TI * NU * 2;
-constexpr int oQhi = 0, oQlo = oQhi + kTile, oK = oQlo + kTile, oV = oK + kKeys, oWhi = oV + kKeys, oWlo = oWhi + kW;
-constexpr int oStage = oWlo + kW;                 // three 32 KB snapshot tiles (kappa hi, kappa lo, nu) leaving by TMA
-constexpr int total = oStage + 3 * kTile + 1024;
-constexpr uint32_t cL = 0, cUk = 64, cUv = 192;
+constexpr int TI = 128, NU = 64, THREADS = 256;
+template <int D> struct Lay {                     // shared-memory offsets and TMEM columns for head dimension D (64 or 128)
+  static constexpr int G = D / 64;                // 64-element (128-byte) column groups of a row
+  static constexpr int kTile = TI * D * 2, kKeys = NU * D * 2, kW = TI * NU * 2;
+  static constexpr int oQhi = 0, oQlo = oQhi + kTile, oK = oQlo + kTile, oV = oK + kKeys, oWhi = oV + kKeys, oWlo = oWhi + kW;
+  static constexpr int oStage = oWlo + kW;        // three snapshot tiles (kappa hi, kappa lo, nu) leaving by TMA
+  static constexpr int total = oStage + 3 * kTile + 1024;
+  static constexpr uint32_t cL = 0, cUk = 64, cUv = 64 + D;
+};
 }  // namespace st
 
 __global__ void k_split_qbar(const float* __restrict__ qbar, long long n, float sigma, bf16* __restrict__ hi, bf16* __restrict__ lo) {
@@ -47,12 +50,17 @@ int split_qbar(const Dims& d, const float* qbar, void* qhi, void* qlo, cudaStrea
   return MUSE_OK;
 }
 
+template <int D>
 __global__ void __launch_bounds__(st::THREADS, 1)
 k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_constant__ CUtensorMap tm_V,
                const __grid_constant__ CUtensorMap tm_okhi, const __grid_constant__ CUtensorMap tm_oklo,
                const __grid_constant__ CUtensorMap tm_onu, const __grid_constant__ CUtensorMap tm_qhi,
                const __grid_constant__ CUtensorMap tm_qlo, const int32_t* __restrict__ off_k, SummPtrs sp, int* __restrict__ status) {
   using namespace st;
+  typedef Lay<D> LY;
+  constexpr int G = LY::G, HD = D / 2, kTile = LY::kTile;
+  constexpr int oQhi = LY::oQhi, oQlo = LY::oQlo, oK = LY::oK, oV = LY::oV, oWhi = LY::oWhi, oWlo = LY::oWlo, oStage = LY::oStage;
+  constexpr uint32_t cL = LY::cL, cUk = LY::cUk, cUv = LY::cUv;
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ uint64_t bar_kv, bar_q, bar1, bar2;
   __shared__ uint32_t tbase_s;
@@ -70,8 +78,10 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
   if (tid == 0) {
     tc::mbar_expect_tx(&bar_q, 2 * kTile);
     const int r = pq * dm.Cq + i0;
-    tc::tma_load_2d(sm + oQhi, &tm_qhi, 0, r, &bar_q); tc::tma_load_2d(sm + oQhi + TI * 128, &tm_qhi, 64, r, &bar_q);
-    tc::tma_load_2d(sm + oQlo, &tm_qlo, 0, r, &bar_q); tc::tma_load_2d(sm + oQlo + TI * 128, &tm_qlo, 64, r, &bar_q);
+    for (int g = 0; g < G; ++g) {
+      tc::tma_load_2d(sm + oQhi + g * TI * 128, &tm_qhi, 64 * g, r, &bar_q);
+      tc::tma_load_2d(sm + oQlo + g * TI * 128, &tm_qlo, 64 * g, r, &bar_q);
+    }
   }
   const uint32_t tbase = tbase_s, tlane = tbase + ((uint32_t)((warp & 3) * 32) << 16);
   const uint32_t aQhi = tc::smem_u32(sm + oQhi), aQlo = tc::smem_u32(sm + oQlo), aK = tc::smem_u32(sm + oK),
@@ -96,12 +106,13 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
   // A bucket usually holds far fewer than 64 keys: only the 16-key groups in use are loaded and contracted.
   auto issue_kv = [&](int c0, int nk) {
     const int ng_ = (nk + 15) >> 4;
-    tc::mbar_expect_tx(&bar_kv, ng_ * 4 * (16 * 128));
+    tc::mbar_expect_tx(&bar_kv, ng_ * 2 * G * (16 * 128));
     const int r = (int)((size_t)pk * dm.N + c0);
-    for (int g = 0; g < ng_; ++g) {
-      tc::tma_load_2d(sm + oK + g * 16 * 128, &tm_K, 0, r + 16 * g, &bar_kv); tc::tma_load_2d(sm + oK + NU * 128 + g * 16 * 128, &tm_K, 64, r + 16 * g, &bar_kv);
-      tc::tma_load_2d(sm + oV + g * 16 * 128, &tm_V, 0, r + 16 * g, &bar_kv); tc::tma_load_2d(sm + oV + NU * 128 + g * 16 * 128, &tm_V, 64, r + 16 * g, &bar_kv);
-    }
+    for (int g = 0; g < ng_; ++g)
+      for (int cg = 0; cg < G; ++cg) {
+        tc::tma_load_2d(sm + oK + cg * NU * 128 + g * 16 * 128, &tm_K, 64 * cg, r + 16 * g, &bar_kv);
+        tc::tma_load_2d(sm + oV + cg * NU * 128 + g * 16 * 128, &tm_V, 64 * cg, r + 16 * g, &bar_kv);
+      }
   };
   auto issue_after = [&](int c_end) {                  // the chunk that starts at key c_end, if any
     int npl = 0;
@@ -191,7 +202,7 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
       if (tid == 32 && ok) issue_after(c0 + nk);         // key / value tiles are free again (not thread 0: it issues the MMAs)
       PCLK(3)
 #pragma unroll
-      for (int d0 = 0; d0 < D; d0 += 32) {              // acc[0..63]: kappa dims 64 wg.., acc[64..127]: nu dims 64 wg..
+      for (int d0 = 0; d0 < D; d0 += 32) {              // acc[0..D/2): kappa dims (D/2) wg.., acc[D/2..D): nu dims (D/2) wg..
         float v[32];
         tc::tmem_ld32(tlane + (d0 < D / 2 ? cUk : cUv) + (D / 2) * wg + (d0 & (D / 2 - 1)), v);
 #pragma unroll
@@ -217,37 +228,33 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
     // by TMA (rows of consecutive query clusters are Ck entries apart in memory) while the next plane is computed
     if (tid == 0) tc::tma_store_wait_read();                           // the previous plane's stores have read the tiles
     __syncthreads();
+    // this warpgroup's half of the row (dims [HD wg, HD wg + HD)) in 16-byte chunks of 8 dims: chunk c of column group gq
 #pragma unroll
-    for (int ck = 0; ck < D / 16; ++ck) {                // this warpgroup's half of the kappa row: hi and lo tiles
-      uint32_t w[4], wl_[4];
+    for (int ck = 0; ck < HD / 8; ++ck) {
+      uint32_t w[4], wl_[4], wn[4];
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const float x0 = acc[ck * 8 + 2 * e] * inv, x1 = acc[ck * 8 + 2 * e + 1] * inv;
         __nv_bfloat162 hh = __floats2bfloat162_rn(x0, x1);
         __nv_bfloat162 ll = __floats2bfloat162_rn(x0 - __low2float(hh), x1 - __high2float(hh));
-        w[e] = *reinterpret_cast<uint32_t*>(&hh); wl_[e] = *reinterpret_cast<uint32_t*>(&ll);
+        __nv_bfloat162 nn = __floats2bfloat162_rn(acc[HD + ck * 8 + 2 * e] * inv, acc[HD + ck * 8 + 2 * e + 1] * inv);
+        w[e] = *reinterpret_cast<uint32_t*>(&hh); wl_[e] = *reinterpret_cast<uint32_t*>(&ll); wn[e] = *reinterpret_cast<uint32_t*>(&nn);
       }
-      const uint32_t off = wg * TI * 128 + tc::sw128_off(row, ck);       // 64-column group wg of the tile
+      const int dch = wg * (HD / 8) + ck;                                  // 16-byte chunk of the whole row
+      const uint32_t off = (dch >> 3) * TI * 128 + tc::sw128_off(row, dch & 7);
       *reinterpret_cast<uint4*>(sm + oStage + off) = make_uint4(w[0], w[1], w[2], w[3]);
       *reinterpret_cast<uint4*>(sm + oStage + kTile + off) = make_uint4(wl_[0], wl_[1], wl_[2], wl_[3]);
-    }
-#pragma unroll
-    for (int ck = 0; ck < D / 16; ++ck) {                // and its half of the nu row
-      uint32_t w[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        __nv_bfloat162 hh = __floats2bfloat162_rn(acc[D / 2 + ck * 8 + 2 * e] * inv, acc[D / 2 + ck * 8 + 2 * e + 1] * inv);
-        w[e] = *reinterpret_cast<uint32_t*>(&hh);
-      }
-      *reinterpret_cast<uint4*>(sm + oStage + 2 * kTile + wg * TI * 128 + tc::sw128_off(row, ck)) = make_uint4(w[0], w[1], w[2], w[3]);
+      *reinterpret_cast<uint4*>(sm + oStage + 2 * kTile + off) = make_uint4(wn[0], wn[1], wn[2], wn[3]);
     }
     tc::fence_async_smem();
     __syncthreads();
     if (tid == 0 && ok) {
       const int P = pq * dm.SB + pl;
-      tc::tma_store_4d(&tm_okhi, sm + oStage, 0, j, i0, P);              tc::tma_store_4d(&tm_okhi, sm + oStage + TI * 128, 64, j, i0, P);
-      tc::tma_store_4d(&tm_oklo, sm + oStage + kTile, 0, j, i0, P);      tc::tma_store_4d(&tm_oklo, sm + oStage + kTile + TI * 128, 64, j, i0, P);
-      tc::tma_store_4d(&tm_onu, sm + oStage + 2 * kTile, 0, j, i0, P);   tc::tma_store_4d(&tm_onu, sm + oStage + 2 * kTile + TI * 128, 64, j, i0, P);
+      for (int g = 0; g < G; ++g) {
+        tc::tma_store_4d(&tm_okhi, sm + oStage + g * TI * 128, 64 * g, j, i0, P);
+        tc::tma_store_4d(&tm_oklo, sm + oStage + kTile + g * TI * 128, 64 * g, j, i0, P);
+        tc::tma_store_4d(&tm_onu, sm + oStage + 2 * kTile + g * TI * 128, 64 * g, j, i0, P);
+      }
       tc::tma_store_commit();
     }
     PCLK(5)
@@ -262,34 +269,40 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
   if (!ok && tid == 0) report_status(status, 7);
 }
 
-bool summarize_tc_supported(const Dims& d, int dtype) { return dtype == MUSE_BF16 && d.D == st::D; }
+bool summarize_tc_supported(const Dims& d, int dtype) { return dtype == MUSE_BF16 && (d.D == 64 || d.D == 128); }
 
 int summarize_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const float* qbar, const SummPtrs& sp,
                  void* qsplit, int* status, cudaStream_t stream) {
   // qsplit: 2 * B*Hq*Cq*D bf16 of scratch for the split centroids
   bf16* qhi = (bf16*)qsplit;
-  bf16* qlo = qhi + (size_t)d.B * d.Hq * d.Cq * st::D;
+  bf16* qlo = qhi + (size_t)d.B * d.Hq * d.Cq * d.D;
   int rcq = split_qbar(d, qbar, qhi, qlo, stream);
   if (rcq != MUSE_OK) return rcq;
   CUtensorMap tqh, tql;
-  rcq = make_tmap_bf16_rows(&tqh, qhi, (uint64_t)d.B * d.Hq * d.Cq, st::D, st::TI);
-  if (rcq == MUSE_OK) rcq = make_tmap_bf16_rows(&tql, qlo, (uint64_t)d.B * d.Hq * d.Cq, st::D, st::TI);
+  rcq = make_tmap_bf16_rows(&tqh, qhi, (uint64_t)d.B * d.Hq * d.Cq, d.D, st::TI);
+  if (rcq == MUSE_OK) rcq = make_tmap_bf16_rows(&tql, qlo, (uint64_t)d.B * d.Hq * d.Cq, d.D, st::TI);
   if (rcq != MUSE_OK) return rcq;
   CUtensorMap tK, tV;
-  int rc = make_tmap_bf16_rows(&tK, Kp, (uint64_t)d.B * d.Hkv * d.N, st::D, 16);       // boxes of 16 keys
-  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tV, Vp, (uint64_t)d.B * d.Hkv * d.N, st::D, 16);
+  int rc = make_tmap_bf16_rows(&tK, Kp, (uint64_t)d.B * d.Hkv * d.N, d.D, 16);       // boxes of 16 keys
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tV, Vp, (uint64_t)d.B * d.Hkv * d.N, d.D, 16);
   // outputs as 4-D tensors (d, j, i, head * planes + plane); a box is 128 query clusters of one key cluster
   CUtensorMap okhi, oklo, onu;
-  const uint64_t dims[4] = {(uint64_t)st::D, (uint64_t)d.Ck, (uint64_t)d.Cq, (uint64_t)d.B * d.Hq * d.SB};
-  const uint64_t strides[3] = {(uint64_t)st::D * 2, (uint64_t)d.Ck * st::D * 2, (uint64_t)d.Cq * d.Ck * st::D * 2};
+  const uint64_t dims[4] = {(uint64_t)d.D, (uint64_t)d.Ck, (uint64_t)d.Cq, (uint64_t)d.B * d.Hq * d.SB};
+  const uint64_t strides[3] = {(uint64_t)d.D * 2, (uint64_t)d.Ck * d.D * 2, (uint64_t)d.Cq * d.Ck * d.D * 2};
   const uint32_t box[4] = {64, 1, (uint32_t)st::TI, 1};
   if (rc == MUSE_OK) rc = make_tmap_bf16_nd(&okhi, sp.khi, 4, dims, strides, box);
   if (rc == MUSE_OK) rc = make_tmap_bf16_nd(&oklo, sp.klo, 4, dims, strides, box);
   if (rc == MUSE_OK) rc = make_tmap_bf16_nd(&onu, sp.nu, 4, dims, strides, box);
   if (rc != MUSE_OK) return rc;
-  MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, st::total));
   prof_mark("k_summarize_tc", stream);
-  k_summarize_tc<<<dim3(d.Ck, cdiv(d.Cq, st::TI), d.B * d.Hq), st::THREADS, st::total, stream>>>(d, tK, tV, okhi, oklo, onu, tqh, tql, off_k, sp, status);
+  const dim3 grid(d.Ck, cdiv(d.Cq, st::TI), d.B * d.Hq);
+  if (d.D == 128) {
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, st::Lay<128>::total));
+    k_summarize_tc<128><<<grid, st::THREADS, st::Lay<128>::total, stream>>>(d, tK, tV, okhi, oklo, onu, tqh, tql, off_k, sp, status);
+  } else {
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, st::Lay<64>::total));
+    k_summarize_tc<64><<<grid, st::THREADS, st::Lay<64>::total, stream>>>(d, tK, tV, okhi, oklo, onu, tqh, tql, off_k, sp, status);
+  }
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }

@@ -66,6 +66,10 @@ WORKLOADS = {
                       rope_theta=5.0e5, student_t_nu=4.0, seed=20250912),
     "headline": Workload("headline", 1, 16, 16, 65536, 128, 256, 1024, 32, components=1024,
                          rope_theta=5.0e5, seed=20250913),
+    # the configuration of the paper's runtime comparison (Section "Experiments", Table 1): 64 heads of
+    # dimension 64, two sequences of 64k tokens, 128 query and 128 key clusters, 8 retrieved clusters, 8k blocks
+    "paper1b": Workload("paper1b", 2, 64, 64, 65536, 64, 128, 128, 8, components=128,
+                        rope_theta=5.0e5, seed=20250915),
     "gqa8b": Workload("gqa8b", 1, 32, 8, 131072, 128, 512, 2048, 32, components=2048,
                       rope_theta=5.0e5, student_t_nu=4.0, outlier_frac=0.01, seed=20250914),
 }

@@ -18,6 +18,8 @@ CASES = {
     "gqa_bf16": wl.WORKLOADS["small"].with_(B=2, Hq=4, Hkv=2, N=2000, Cq=16, Ck=40, m=6, components=64),
     "d128": wl.WORKLOADS["headline"].with_(Hq=2, Hkv=1, N=3072, Cq=24, Ck=128, m=8, components=96),
     "d128_wide": wl.WORKLOADS["headline"].with_(name="headline_wide", Hq=1, Hkv=1, N=2048, Cq=4, Ck=256, m=16, components=64),
+    # D = 64 with C_k a multiple of 128: the shapes at which the D = 64 instances of the tensor-core far-field kernels run
+    "d64": wl.WORKLOADS["small"].with_(name="small_d64", B=1, Hq=2, Hkv=1, N=3072, Cq=24, Ck=128, m=8, components=96),
 }
 
 

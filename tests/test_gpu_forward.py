@@ -81,6 +81,8 @@ def test_summaries_match_oracle(name, gain):
 TC = {
     "tc": CASES["d128"].with_(name="tc", Hq=2, Hkv=1, N=4096, S=4, Cq=16, Ck=256, m=4),
     "tc_gqa4": CASES["d128"].with_(name="tc_gqa4", Hq=4, Hkv=1, N=2048, S=4, Cq=8, Ck=128, m=4),
+    "tc_d64": CASES["d64"].with_(name="tc_d64", Hq=2, Hkv=1, N=4096, S=4, Cq=16, Ck=256, m=4),
+    "tc_d64_gqa4": CASES["d64"].with_(name="tc_d64_gqa4", Hq=4, Hkv=1, N=2048, S=4, Cq=8, Ck=128, m=4),
 }
 TC_FWD_KERNELS = {"k_summarize_tc", "k_far_fwd_tc", "k_local_fwd_tc"}
 TC_BWD_KERNELS = {"k_far_bwd_tc", "k_summ_bwd_tc"}
