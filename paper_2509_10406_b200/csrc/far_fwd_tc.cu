@@ -24,7 +24,6 @@ constexpr int kFJ = 128;                            // clusters per tile
 // Queries per pass FR and per selection step FQ (one warp each) are template parameters: 64 / 16 up to 1024
 // key clusters, 32 / 8 up to 2048 (all FR x Ck scores of a pass live in the 512 TMEM columns, P and the score
 // rows of a step in shared memory).
-constexpr int kFarTcCols = 512;
 constexpr int kMaxStA = 6, kMaxStD = 4;
 constexpr int kCandMax = 128;                       // candidates kept by the compacting selection (4 per lane)
 
@@ -221,13 +220,16 @@ __device__ __forceinline__ void select_top_m(float* s, int Ck, int m, int32_t* s
   for (int k = base + lane; k < m; k += 32) so[k] = -1;
 }
 
-template <int FR, int FQ, int D>
-__global__ void __launch_bounds__(FQ * 32, 1)
+// NKMAX: scores per lane that the selection keeps in registers (Ck <= 32 NKMAX); MINB: CTAs per SM the register
+// budget is set for.  With few key clusters the per-query selection, a chain of dependent warp operations, is what
+// takes the time: small instances (few registers, few TMEM columns) put several CTAs on an SM.
+template <int FR, int FQ, int D, int NKMAX, int MINB>
+__global__ void __launch_bounds__(FQ * 32, MINB)
 k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_constant__ CUtensorMap tm_klo,
              const __grid_constant__ CUtensorMap tm_nu, const bf16* __restrict__ Q, const int32_t* __restrict__ off_q,
              const int32_t* __restrict__ perm_q, const float* __restrict__ mu, const float* __restrict__ beta,
              const int32_t* __restrict__ sel_in, int32_t* __restrict__ sel_out, float* __restrict__ o_far,
-             float* __restrict__ lse_far, int p_bytes, int sc_bytes, int nsA, int nsD, int* __restrict__ status) {
+             float* __restrict__ lse_far, int p_bytes, int sc_bytes, int nsA, int nsD, int tcols, int* __restrict__ status) {
   constexpr int NT = FQ * 32, NTG = FQ / 4, KT = 16 / NTG;   // threads; tile groups in the TMEM read-out; cluster tiles per group
   constexpr int kTileBytes = kFJ * D * 2, G = D / 64;        // one [128 clusters][D] bf16 operand tile; 128-byte column groups of a row
   extern __shared__ __align__(1024) unsigned char sm_raw[];
@@ -254,7 +256,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   const bf16* Qp = Q + (size_t)pq * dm.N * D;
   const int32_t* pm = perm_q + (size_t)pq * dm.N;
 
-  if (warp == 0) tc::tmem_alloc(&tbase_s, kFarTcCols);
+  if (warp == 0) tc::tmem_alloc(&tbase_s, tcols);
   if (tid == 0) {
     for (int s = 0; s < kMaxStA; ++s) { tc::mbar_init(&bars.fullA[s], 1); tc::mbar_init(&bars.emptyA[s], 1); }
     for (int s = 0; s < kMaxStD; ++s) { tc::mbar_init(&bars.fullD[s], 1); tc::mbar_init(&bars.emptyD[s], 1); }
@@ -423,7 +425,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #ifdef MUSE_PHASE_CLOCKS
           if (warp == 0 && blockIdx.x == 200 && blockIdx.y == 5 && blockIdx.z == 1 && r0 == p0 && qs == 0) dbg = status + 56;
 #endif
-          select_top_m<(FR == 64 ? 32 : 64)>(s, Ck, m, so, lane, Pm + r * 128, FR * 128, Ck >= 512, dbg);
+          select_top_m<NKMAX>(s, Ck, m, so, lane, Pm + r * 128, FR * 128, Ck >= 512, dbg);
         }
         __syncwarp();
 #ifdef MUSE_PHASE_CLOCKS
@@ -538,7 +540,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
   }
   tc::fence_before_sync();
   __syncthreads();
-  if (warp == 0) tc::tmem_dealloc(tbase, kFarTcCols);
+  if (warp == 0) tc::tmem_dealloc(tbase, tcols);
   if (!ok && tid == 0) report_status(status, 3);
 }
 
@@ -566,14 +568,18 @@ int far_fwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const int32_t* 
   // (D = 64: one more tile of room behind the ring, which the padded 128-row products of phase D read past)
   const size_t smem = (size_t)p_bytes + sc_bytes + FR * d.D * 2 + 1024 + (d.D == 64 ? tile_bytes : 0);
   prof_mark("k_far_fwd_tc", st);
-#define MUSE_FAR_FWD_LAUNCH(FR_, FQ_, D_)                                                                                   \
-  do {                                                                                                                    \
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_fwd_tc<FR_, FQ_, D_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-    k_far_fwd_tc<FR_, FQ_, D_><<<dim3(d.Cq, d.SB, d.B * d.Hq), FQ_ * 32, smem, st>>>(                                       \
-        d, khi, klo, nu, (const bf16*)Q, off_q, perm_q, sp.mu, sp.beta, sel_in, sel_out, o_far, lse_far, p_bytes, sc_bytes, nsA, nsD, status); \
+  // TMEM columns: all FR x Ck scores of a pass (the output of phase D reuses them), a power of two >= 32
+  int tcols = 32;
+  while (tcols < FR * (d.Ck / kFJ)) tcols *= 2;
+#define MUSE_FAR_FWD_LAUNCH(FR_, FQ_, D_, NK_, MB_)                                                                              \
+  do {                                                                                                                         \
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_fwd_tc<FR_, FQ_, D_, NK_, MB_>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+    k_far_fwd_tc<FR_, FQ_, D_, NK_, MB_><<<dim3(d.Cq, d.SB, d.B * d.Hq), FQ_ * 32, smem, st>>>(                                   \
+        d, khi, klo, nu, (const bf16*)Q, off_q, perm_q, sp.mu, sp.beta, sel_in, sel_out, o_far, lse_far, p_bytes, sc_bytes, nsA, nsD, tcols, status); \
   } while (0)
-  if (wide) { if (d.D == 128) MUSE_FAR_FWD_LAUNCH(32, 8, 128); else MUSE_FAR_FWD_LAUNCH(32, 8, 64); }
-  else { if (d.D == 128) MUSE_FAR_FWD_LAUNCH(64, 16, 128); else MUSE_FAR_FWD_LAUNCH(64, 16, 64); }
+  if (wide) { if (d.D == 128) MUSE_FAR_FWD_LAUNCH(32, 8, 128, 64, 1); else MUSE_FAR_FWD_LAUNCH(32, 8, 64, 64, 1); }
+  else if (d.Ck <= 256) { if (d.D == 128) MUSE_FAR_FWD_LAUNCH(64, 16, 128, 8, 2); else MUSE_FAR_FWD_LAUNCH(64, 16, 64, 8, 2); }
+  else { if (d.D == 128) MUSE_FAR_FWD_LAUNCH(64, 16, 128, 32, 1); else MUSE_FAR_FWD_LAUNCH(64, 16, 64, 32, 1); }
 #undef MUSE_FAR_FWD_LAUNCH
   MUSE_LAUNCH_OK();
   return MUSE_OK;

@@ -1,5 +1,5 @@
 // Exact retrieval, backward (Section "Exact Retrieval and Local Attention"; gradients with the selections
-// held constant, Appendix "Centroid Gradient Flow"), D = 128.  With L the merged log-sum-exp and
+// held constant, Appendix "Centroid Gradient Flow"), D = 64 or 128.  With L the merged log-sum-exp and
 // delta = dO.O:   P = exp(sigma q.k - L),  G = sigma P (dO.v - delta),
 //                 dQ = G K  (one bf16 partial row per (query, slot) pair),  dV = P^T dO,  dK = G^T Q.
 // Organised by the inverse index like the forward pass: a CTA owns one key cluster of one head (or a share
@@ -26,14 +26,16 @@ namespace muse {
 typedef __nv_bfloat16 bf16;
 
 namespace rb {
-constexpr int D = 128, kPairs = 128, kKeys = 64;
+constexpr int kPairs = 128, kKeys = 64;
 constexpr int kRowWarps = 4, kIssuerWarp0 = 8, kGatherWarp0 = 10, kGather = 128, kThreads = (kGatherWarp0 + 2 * kGather / 32) * 32;
 constexpr int kSplit = 4, kTilesPerCta = 16;                // a cluster with many pair tiles is shared by up to 4 CTAs
 constexpr int kOkCache = 72;
 constexpr float kLog2e = 1.4426950408889634f;
-constexpr int kTile = kPairs * D * 2, kKV = kKeys * D * 2, kPG = kPairs * kKeys * 2;
-constexpr int oK = 0, oV = kKV, oHalf = 2 * kKV, kHalf = 2 * kTile + 2 * kPG;   // per half: Q | dO | P | G
-constexpr int kSmem = oHalf + 2 * kHalf;                    // 224 KB: no slack, the kernel checks the alignment of its base
+template <int D> struct Lay {
+  static constexpr int kTile = kPairs * D * 2, kKV = kKeys * D * 2, kPG = kPairs * kKeys * 2;
+  static constexpr int oK = 0, oV = kKV, oHalf = 2 * kKV, kHalf = 2 * kTile + 2 * kPG;   // per half: Q | dO | P | G
+  static constexpr int kSmem = oHalf + 2 * kHalf;           // 224 KB at D = 128: no slack, the kernel checks the alignment of its base
+};
 constexpr uint32_t cS = 0, cDP = 64, cDQ = 0, cDV = 128, cDK = 192, kCols = 256;   // per half; dQ reuses the columns of S and dP
 
 struct Bars { uint64_t q_full, q_empty, s_done, pg_ready, m2_done, dq_free; };
@@ -51,12 +53,15 @@ template <int ROWS> __device__ __forceinline__ uint64_t desc_mn(uint32_t base, i
 }
 }  // namespace rb
 
+template <int D>
 __global__ void __launch_bounds__(rb::kThreads, 1)
 k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ dO, const bf16* __restrict__ Kp,
                    const bf16* __restrict__ Vp, const float* __restrict__ LSE, const float* __restrict__ delta,
                    const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
                    bf16* __restrict__ dq_part, float* __restrict__ dK_perm, float* __restrict__ dV_perm, int* __restrict__ status) {
   using namespace rb;
+  typedef Lay<D> LY;
+  constexpr int kTile = LY::kTile, kPG = LY::kPG, oK = LY::oK, oV = LY::oV, oHalf = LY::oHalf, kHalf = LY::kHalf;
   extern __shared__ __align__(1024) unsigned char sm[];
   __shared__ Bars bars[2];
   __shared__ uint32_t tbase_s;
@@ -248,7 +253,7 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       }
       // dV^T and dK^T of this sweep's keys: thread = output dim, one key per column; the other half of the CTA
       // (and other CTAs that share the cluster) add theirs to the same rows
-      if (started) {
+      if (started && (warp & 3) * 32 < D) {                  // (warp-uniform: the lanes of a warp hold 32 consecutive dims)
         const int dd = (warp & 3) * 32 + lane;
 #pragma unroll
         for (int w2 = 0; w2 < 2; ++w2) {
@@ -290,7 +295,9 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
           tc::fence_after_sync();
           RBCLK(4)
           const uint32_t id_dq = tc::idesc_bf16(kPairs, D, 0, 1);        // A = G (contraction over keys), B = key rows MN-major
-          const uint32_t id_t = tc::idesc_bf16(D, kKeys, 1, 1);          // A = dO / Q tile and B = P / G tile, both contracted over pairs
+          // A = dO / Q tile and B = P / G tile, both contracted over pairs.  M = 128 output dims even when D = 64: the second
+          // 64-dim group of the A operand is then the tile that follows in shared memory, and lanes 64..127 hold numbers nobody reads
+          const uint32_t id_t = tc::idesc_bf16(128, kKeys, 1, 1);
           const bool acc = np > np0;                                     // the accumulators start at zero in every sweep
 #pragma unroll
           for (int ks = 0; ks < kKeys / 16; ++ks)
@@ -376,10 +383,17 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
 int ret_bwd_pairs_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, const void* Vp, const float* LSE,
                      const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, void* dq_part,
                      float* dK_perm, float* dV_perm, int* status, cudaStream_t st) {
-  MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_bwd_pairs_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, rb::kSmem));
   prof_mark("k_ret_bwd_pairs_tc", st);
-  k_ret_bwd_pairs_tc<<<dim3(d.Ck, rb::kSplit, d.B * d.Hq), rb::kThreads, rb::kSmem, st>>>(
-      d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp, (const bf16*)Vp, LSE, delta, off_k, goff, pairs, (bf16*)dq_part, dK_perm, dV_perm, status);
+  const dim3 grid(d.Ck, rb::kSplit, d.B * d.Hq);
+  if (d.D == 128) {
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_bwd_pairs_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, rb::Lay<128>::kSmem));
+    k_ret_bwd_pairs_tc<128><<<grid, rb::kThreads, rb::Lay<128>::kSmem, st>>>(
+        d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp, (const bf16*)Vp, LSE, delta, off_k, goff, pairs, (bf16*)dq_part, dK_perm, dV_perm, status);
+  } else {
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_bwd_pairs_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, rb::Lay<64>::kSmem));
+    k_ret_bwd_pairs_tc<64><<<grid, rb::kThreads, rb::Lay<64>::kSmem, st>>>(
+        d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp, (const bf16*)Vp, LSE, delta, off_k, goff, pairs, (bf16*)dq_part, dK_perm, dV_perm, status);
+  }
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }
