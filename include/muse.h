@@ -88,7 +88,10 @@ typedef struct muse_params {
   int32_t Cq, Ck, m;            /* 1 <= Cq <= 4096, 1 <= Ck <= 4096, 0 <= m <= min(Ck,64)          */
   int32_t causal;               /* 1: blocked causal handling of the paper; 0: one block, no local */
   int32_t n_blocks;             /* S, spatial blocks (0 -> 8); N % S == 0; forced to 1 if !causal  */
-  int32_t k2;                   /* spatial selection: 0 = all visible blocks (the only value built) */
+  int32_t k2;                   /* spatial selection inside the selected clusters (Section "Two-Level Retrieval"):
+                                   0 = every earlier block is retrieved; 1..8 = only the k2 best-scoring earlier
+                                   blocks, the others enter through their per-block summaries (bf16 mode, causal,
+                                   forward only; ignored when !causal)                                           */
   int32_t dtype;                /* MUSE_BF16 | MUSE_F32: type of Q,K,V,O,dO,dQ,dK,dV               */
   float   softmax_scale;        /* sigma; <= 0 -> 1/sqrt(D)                                        */
   int32_t kmeans_iters;         /* T Lloyd iterations before the final assignment (>= 0)           */
@@ -124,8 +127,12 @@ MUSE_API int muse_workspace_bytes(const muse_params_t* p, size_t out[6]);
  *   off[5], off[6]          K and V bucketed by (cluster, block), [B,Hkv,N,D] dtype
  *   off[7] cbar             dipole == 1 only: merged dipole matrices Cbar = sum_j p(j) Cov_0j(v,k),
  *                           [B,Hq,SB,Cq][D value dims][D key dims], fp32 (fp32 mode) or bf16; with
- *                           dipole == 0 nothing is stored there (off[7] = end of the buffer) */
-MUSE_API int muse_summaries_layout(const muse_params_t* p, size_t off[8]);
+ *                           dipole == 0 nothing is stored there
+ *   off[8] per-block set    k2 > 0 only: a second mu | beta | kappa | kappa_lo | nu group of the same shapes
+ *                           and spacing as off[0..4], holding the summaries of each block alone (plane s =
+ *                           the keys of block s), which the spatial block selection scores; with k2 == 0
+ *                           nothing is stored there (off[8] = end of the buffer) */
+MUSE_API int muse_summaries_layout(const muse_params_t* p, size_t off[9]);
 
 /* Lloyd k-means of the queries (per query head, Cq clusters) and keys (per kv head, Ck
  * clusters): T x (assign to argmin_c |c|^2 - 2 x.c, lowest index on ties; move each centre to
@@ -193,14 +200,18 @@ MUSE_API int muse_summarize(const muse_params_t* p, const void* K, const void* V
  * attention, approximate the rest with the summaries, add exact causal attention inside the
  * query's block, merge by log-sum-exp.
  *   sel_in   in   [B,Hq,N,m] clusters to retrieve (-1 = none) or NULL to select here
+ *   bsel_in  in   k2 > 0: [B,Hq,N,m,k2] blocks to retrieve inside each selected cluster (-1 = none), in
+ *                 the slot order of sel_in, or NULL to select here; ignored when k2 == 0
  *   O        out  [B,Hq,N,D] dtype
  *   LSE      out  [B,Hq,N] fp32 log of the merged normaliser
- *   sel_out  out  [B,Hq,N,m] retrieved clusters in no particular order, padded with -1 (may be NULL) */
+ *   sel_out  out  [B,Hq,N,m] retrieved clusters in no particular order, padded with -1 (may be NULL)
+ *   bsel_out out  k2 > 0: [B,Hq,N,m,k2] retrieved blocks of each slot of sel_out, best first, -1 padded
+ *                 (may be NULL) */
 MUSE_API int muse_attn_fwd(const muse_params_t* p, const void* Q, const void* K, const void* V,
                   const int32_t* assign_q, const float* qbar,
                   const int32_t* off_k, const int32_t* perm_k, const void* summaries,
-                  const int32_t* sel_in, void* O, float* LSE, int32_t* sel_out,
-                  void* ws, size_t ws_bytes, cudaStream_t stream);
+                  const int32_t* sel_in, const int32_t* bsel_in, void* O, float* LSE, int32_t* sel_out,
+                  int32_t* bsel_out, void* ws, size_t ws_bytes, cudaStream_t stream);
 
 /* Backward of sum(O * dO) w.r.t. Q, K, V with assign_*, sel and qbar constant; dK, dV of a
  * kv head are summed over the query heads that share it.

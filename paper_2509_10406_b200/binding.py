@@ -86,7 +86,7 @@ def lib() -> ctypes.CDLL:
         L.muse_summaries_layout.argtypes = [pp, ctypes.POINTER(sz)]
         L.muse_cluster.argtypes = [pp, vp, vp, i32p, i32p, i32p, i32p, f32p, f32p, vp, sz, vp]
         L.muse_summarize.argtypes = [pp, vp, vp, i32p, f32p, i32p, i32p, i32p, f32p, f32p, vp, vp, sz, vp]
-        L.muse_attn_fwd.argtypes = [pp, vp, vp, vp, i32p, f32p, i32p, i32p, vp, i32p, vp, f32p, i32p, vp, sz, vp]
+        L.muse_attn_fwd.argtypes = [pp, vp, vp, vp, i32p, f32p, i32p, i32p, vp, i32p, i32p, vp, f32p, i32p, i32p, vp, sz, vp]
         L.muse_attn_bwd.argtypes = [pp, vp, vp, vp, vp, f32p, vp, i32p, f32p, i32p, i32p, vp, i32p, vp, vp, vp,
                                     vp, sz, vp]
         L.muse_cluster_noalloc.argtypes = [pp, vp, vp, i32p, i32p, i32p, i32p, f32p, f32p, vp]
@@ -150,8 +150,8 @@ def muse_profile_report() -> dict:
 
 
 def muse_summaries_layout(p: MuseParams):
-    """Byte offsets (mu, beta, kappa, kappa_lo, nu, K bucketed, V bucketed)."""
-    out = (ctypes.c_size_t * 8)()
+    """Byte offsets (mu, beta, kappa, kappa_lo, nu, K bucketed, V bucketed, dipole matrices, per-block set)."""
+    out = (ctypes.c_size_t * 9)()
     _check(lib().muse_summaries_layout(ctypes.byref(p), out), "muse_summaries_layout")
     return tuple(int(x) for x in out)
 
@@ -203,10 +203,11 @@ def muse_test_wait_timeout(ws, limit_clocks: int) -> None:
     _check(lib().muse_test_wait_timeout(_ptr(ws), int(limit_clocks), _stream()), "muse_test_wait_timeout")
 
 
-def muse_attn_fwd(p, Q, K, V, assign_q, qbar, off_k, perm_k, summaries, sel_in, O, LSE, sel_out, ws):
+def muse_attn_fwd(p, Q, K, V, assign_q, qbar, off_k, perm_k, summaries, sel_in, O, LSE, sel_out, ws, bsel_in=None,
+                  bsel_out=None):
     _check(lib().muse_attn_fwd(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(assign_q), _ptr(qbar), _ptr(off_k),
-                               _ptr(perm_k), _ptr(summaries), _ptr(sel_in), _ptr(O), _ptr(LSE), _ptr(sel_out),
-                               _ptr(ws), ws.numel() * ws.element_size(), _stream()), "muse_attn_fwd")
+                               _ptr(perm_k), _ptr(summaries), _ptr(sel_in), _ptr(bsel_in), _ptr(O), _ptr(LSE), _ptr(sel_out),
+                               _ptr(bsel_out), _ptr(ws), ws.numel() * ws.element_size(), _stream()), "muse_attn_fwd")
 
 
 def muse_attn_bwd(p, Q, K, V, O, LSE, dO, assign_q, qbar, off_k, perm_k, summaries, sel, dQ, dK, dV, ws):
@@ -236,6 +237,7 @@ class MuseBuffers:
         self.summaries = e(sizes[4], dtype=torch.uint8)
         self.O = e(B, Hq, N, D, dtype=dt); self.LSE = e(B, Hq, N, dtype=f32)
         self.sel = e(B, Hq, N, max(m, 1), dtype=i32)
+        self.bsel = e(B, Hq, N, max(m, 1), max(p.k2, 1), dtype=i32) if p.k2 > 0 else None
         need = max(sizes[:3] + ((sizes[3],) if backward else ()))
         self.sizes = sizes
         self.ws = e(need, dtype=torch.uint8)
@@ -264,7 +266,7 @@ def muse_layer_forward(p, buf: MuseBuffers, Q, K, V, init_q=None, init_k=None, s
     muse_cluster(p, Q, K, init_q, init_k, buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, buf.ws)
     muse_summarize(p, K, V, buf.assign_k, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
     muse_attn_fwd(p, Q, K, V, buf.assign_q, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, sel_in, buf.O, buf.LSE,
-                  buf.sel, buf.ws)
+                  buf.sel, buf.ws, bsel_out=buf.bsel)
     return buf.O
 
 

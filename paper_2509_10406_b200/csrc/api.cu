@@ -37,7 +37,7 @@ int resolve(const muse_params_t* p, Dims* d) {
   if (p->D != 64 && p->D != 128) return MUSE_ERR_UNSUPPORTED;
   if (p->Hq > kMaxHeads || p->m > kMaxM || p->Cq > kMaxC || p->Ck > kMaxC) return MUSE_ERR_UNSUPPORTED;
   if (p->dipole != 0 && p->dipole != 1) return MUSE_ERR_INVALID_ARG;
-  if (p->k2 != 0) return MUSE_ERR_UNSUPPORTED;
+  if (p->k2 > 8 || (p->k2 > 0 && p->dipole != 0)) return MUSE_ERR_UNSUPPORTED;
   if (p->dipole != 0 && p->m != 0) return MUSE_ERR_UNSUPPORTED;      // the paper defines the dipole without retrieval
   int S = p->causal ? (p->n_blocks == 0 ? 8 : p->n_blocks) : 1;
   if (p->N % S != 0) return MUSE_ERR_INVALID_ARG;
@@ -48,6 +48,9 @@ int resolve(const muse_params_t* p, Dims* d) {
   d->S = S; d->SB = p->causal ? S - 1 : 1; d->Bs = p->N / S;
   d->causal = p->causal ? 1 : 0; d->sel_mode = p->sel_mode; d->agg_grad = p->agg_grad ? 1 : 0;
   d->dipole = p->dipole;
+  d->k2 = p->causal ? p->k2 : 0;                          // spatial selection needs spatial blocks
+  if (d->k2 > 0 && S - 1 > 32) return MUSE_ERR_UNSUPPORTED;
+  if (d->k2 > 0 && p->dtype != MUSE_BF16) return MUSE_ERR_UNSUPPORTED;   // built on the bf16 retrieval kernel
   d->sigma = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->D);
   for (int h = 0; h < kMaxHeads; ++h) d->hm.g[h] = 0;
   for (int h = 0; h < p->Hq; ++h) {
@@ -110,13 +113,13 @@ int muse_workspace_bytes(const muse_params_t* p, size_t out[6]) {
   return MUSE_OK;
 }
 
-int muse_summaries_layout(const muse_params_t* p, size_t off[8]) {
+int muse_summaries_layout(const muse_params_t* p, size_t off[9]) {
   Dims d;
   int rc = resolve(p, &d);
   if (rc != MUSE_OK) return rc;
   if (off == nullptr) return MUSE_ERR_INVALID_ARG;
   SummLayout L = summ_layout(d, p->dtype);
-  off[0] = L.mu; off[1] = L.beta; off[2] = L.khi; off[3] = L.klo; off[4] = L.nu; off[5] = L.Kp; off[6] = L.Vp; off[7] = L.cbar;
+  off[0] = L.mu; off[1] = L.beta; off[2] = L.khi; off[3] = L.klo; off[4] = L.nu; off[5] = L.Kp; off[6] = L.Vp; off[7] = L.cbar; off[8] = L.blk;
   return MUSE_OK;
 }
 
@@ -170,8 +173,8 @@ int muse_summarize(const muse_params_t* p, const void* K, const void* V, const i
 
 int muse_attn_fwd(const muse_params_t* p, const void* Q, const void* K, const void* V,
                   const int32_t* assign_q, const float* qbar, const int32_t* off_k, const int32_t* perm_k,
-                  const void* summaries, const int32_t* sel_in, void* O, float* LSE, int32_t* sel_out,
-                  void* ws, size_t ws_bytes, cudaStream_t stream) {
+                  const void* summaries, const int32_t* sel_in, const int32_t* bsel_in, void* O, float* LSE, int32_t* sel_out,
+                  int32_t* bsel_out, void* ws, size_t ws_bytes, cudaStream_t stream) {
   Dims d;
   int rc = resolve(p, &d);
   if (rc != MUSE_OK) return rc;
@@ -181,7 +184,7 @@ int muse_attn_fwd(const muse_params_t* p, const void* Q, const void* K, const vo
   muse_workspace_bytes(p, need);
   if (ws_bytes < need[2]) return MUSE_ERR_WORKSPACE;
   if (clear_status(ws, stream) != MUSE_OK) return MUSE_ERR_CUDA;
-  rc = attn_fwd(d, p->dtype, Q, K, V, assign_q, qbar, off_k, perm_k, summaries, sel_in, O, LSE, sel_out, ws, stream);
+  rc = attn_fwd(d, p->dtype, Q, K, V, assign_q, qbar, off_k, perm_k, summaries, sel_in, bsel_in, O, LSE, sel_out, bsel_out, ws, stream);
   prof_mark(nullptr, stream);
   return rc;
 }
@@ -195,6 +198,7 @@ int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K, const vo
   if (rc != MUSE_OK) return rc;
   if (!Q || !K || !V || !O || !LSE || !dO || !assign_q || !qbar || !off_k || !perm_k || !dQ || !dK || !dV || !ws) return MUSE_ERR_INVALID_ARG;
   if (d.dipole) return MUSE_ERR_UNSUPPORTED;       // no backward through the dipole correction
+  if (d.k2 > 0) return MUSE_ERR_UNSUPPORTED;       // nor, yet, through the spatial block selection (forward only)
   if (d.m > 0 && d.SB > 0 && sel == nullptr) return MUSE_ERR_INVALID_ARG;
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(qbar) ||
       !aligned16(summaries) || !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;

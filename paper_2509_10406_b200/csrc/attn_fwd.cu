@@ -14,7 +14,9 @@ bool far_fwd_tc_supported(const Dims& d, int dtype);
 int far_fwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const int32_t* off_q, const int32_t* perm_q,
                const int32_t* sel_in, int32_t* sel_out, float* o_far, float* lse_far, int* status, cudaStream_t st);
 int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
-               const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st);
+               const int32_t* pairs, const int32_t* bsel, void* o_part, float* l_part, int* status, cudaStream_t st);
+int block_select(const Dims& d, int dtype, const void* Q, const int32_t* assign_q, const int32_t* sel, const SummPtrs& sp,
+                 const int32_t* bsel_in, int32_t* bsel_out, float* o_near, float* lse_near, cudaStream_t st);
 
 // plane of a query = index of the accumulated-summary plane it reads: block - 1 when causal
 // (block 0 sees no far field), 0 when non-causal.
@@ -443,6 +445,7 @@ template <class T, int D, class PT>      // PT: element type of the retrieval pa
 __global__ void k_merge(Dims dm, const float* __restrict__ o_far, const float* __restrict__ lse_far,
                         const float* __restrict__ o_loc, const float* __restrict__ lse_loc,
                         const PT* __restrict__ o_part, const float* __restrict__ l_part,
+                        const float* __restrict__ o_near, const float* __restrict__ lse_near,
                         const int32_t* __restrict__ sel, T* __restrict__ O, float* __restrict__ LSE) {
   const int pq = blockIdx.y;
   const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
@@ -452,7 +455,9 @@ __global__ void k_merge(Dims dm, const float* __restrict__ o_far, const float* _
   const bool far_ok = pl >= 0 && dm.SB > 0;
   const float lf = far_ok ? lse_far[row] : -INFINITY;
   const float ll = dm.causal ? lse_loc[row] : -INFINITY;
-  float mx = fmaxf(lf, ll);
+  // near field (component 2 of the merge): non-retrieved earlier blocks of the selected clusters; empty unless k2 > 0
+  const float ln = (far_ok && lse_near != nullptr) ? lse_near[row] : -INFINITY;
+  float mx = fmaxf(fmaxf(lf, ll), ln);
   const int m = dm.m;
   float lp_mine[2] = {-INFINITY, -INFINITY};        // slots lane, lane + 32
   if (far_ok) {
@@ -469,7 +474,8 @@ __global__ void k_merge(Dims dm, const float* __restrict__ o_far, const float* _
   for (int a = 0; a < 2; ++a) tot += lp_mine[a] == -INFINITY ? 0.f : expf(lp_mine[a] - mx);
   tot = warp_sum(tot);
   const float wf = lf == -INFINITY ? 0.f : expf(lf - mx), wl = ll == -INFINITY ? 0.f : expf(ll - mx);
-  tot += wf + wl;
+  const float wn = ln == -INFINITY ? 0.f : expf(ln - mx);
+  tot += wf + wl + wn;
   const float inv = 1.f / tot;
   // lane owns EPL consecutive output dims: one vector load per input row and lane
   constexpr int EPL = D / 32;
@@ -488,6 +494,12 @@ __global__ void k_merge(Dims dm, const float* __restrict__ o_far, const float* _
     ldv<EPL>(o_loc + row * D + dd, x);
 #pragma unroll
     for (int k = 0; k < EPL; ++k) acc[k] = fmaf(wl, x[k], acc[k]);
+  }
+  if (wn > 0.f) {
+    float x[EPL];
+    ldv<EPL>(o_near + row * D + dd, x);
+#pragma unroll
+    for (int k = 0; k < EPL; ++k) acc[k] = fmaf(wn, x[k], acc[k]);
   }
   // retrieved slots four at a time, so that four independent row loads are in flight
   for (int s0 = 0; s0 < m; s0 += 4) {
@@ -515,7 +527,9 @@ __global__ void k_merge(Dims dm, const float* __restrict__ o_far, const float* _
 }
 
 // ---------------------------------------------------------------------------------------------
-struct FwdWs { int32_t *status, *off_q, *perm_q, *sort_scratch, *ret_scratch, *sel_tmp; float *o_far, *lse_far, *o_loc, *lse_loc, *o_part, *l_part; };
+template <class T> constexpr bool kTensorT() { return sizeof(T) == 2; }
+
+struct FwdWs { int32_t *status, *off_q, *perm_q, *sort_scratch, *ret_scratch, *sel_tmp, *bsel_tmp; float *o_far, *lse_far, *o_loc, *lse_loc, *o_part, *l_part, *o_near, *lse_near; };
 
 static FwdWs fwd_ws(const Dims& d, Arena& ar) {
   FwdWs w;
@@ -532,6 +546,10 @@ static FwdWs fwd_ws(const Dims& d, Arena& ar) {
   w.lse_loc = ar.take<float>(pq * d.N);
   w.o_part = ar.take<float>(pq * d.N * d.m * d.D);
   w.l_part = ar.take<float>(pq * d.N * d.m);
+  const bool two_level = d.k2 > 0 && d.causal;
+  w.bsel_tmp = ar.take<int32_t>(two_level ? pq * d.N * d.m * d.k2 : 0);
+  w.o_near = ar.take<float>(two_level ? pq * d.N * d.D : 0);
+  w.lse_near = ar.take<float>(two_level ? pq * d.N : 0);
   return w;
 }
 
@@ -540,7 +558,8 @@ size_t attn_fwd_ws_bytes(const Dims& d, int) { Arena ar(nullptr); fwd_ws(d, ar);
 template <class T, int D>
 static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const int32_t* assign_q,
                       const float* qbar, const int32_t* off_k, const int32_t* perm_k, const void* summaries,
-                      const int32_t* sel_in, T* O, float* LSE, int32_t* sel_out, void* ws, int dtype, cudaStream_t st) {
+                      const int32_t* sel_in, const int32_t* bsel_in, T* O, float* LSE, int32_t* sel_out, int32_t* bsel_out, void* ws,
+                      int dtype, cudaStream_t st) {
   Arena ar(ws);
   FwdWs w = fwd_ws(d, ar);
   const int pq = d.B * d.Hq;
@@ -548,6 +567,9 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
   const char* base = (const char*)summaries;
   const T* Kp = (const T*)(base + L.Kp); const T* Vp = (const T*)(base + L.Vp);
   int32_t* sel = sel_out ? sel_out : w.sel_tmp;
+  const bool two_level = d.k2 > 0 && d.causal && d.m > 0;
+  int32_t* bsel = two_level ? (bsel_out ? bsel_out : w.bsel_tmp) : nullptr;
+  if (two_level && !kTensorT<T>()) return MUSE_ERR_UNSUPPORTED;   // spatial block selection is built on the bf16 retrieval kernel
   const size_t fl_smem = 3 * tile_bytes<T, D>() + ptile_bytes();
   constexpr bool kTensor = sizeof(T) == 2;      // bf16 mode runs the exact-attention parts on tcgen05
   // local attention
@@ -581,12 +603,17 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
       rc = dipole_apply(d, dtype, Q, qbar, w.off_q, w.perm_q, base + L.cbar, w.lse_far, w.o_far, st);
       if (rc != MUSE_OK) return rc;
     }
+    if (two_level) {
+      // second level: the k2 best earlier blocks of every selected cluster, and the near field of the others
+      rc = block_select(d, dtype, Q, assign_q, sel, summ_ptrs_blk(L, base), bsel_in, bsel, w.o_near, w.lse_near, st);
+      if (rc != MUSE_OK) return rc;
+    }
     if (d.m > 0) {
       RetIndex ri;
       rc = build_ret_index(d, sel, w.ret_scratch, &ri, st);
       if (rc != MUSE_OK) return rc;
       if (kTensor) {
-        rc = ret_fwd_tc(d, Q, Kp, Vp, off_k, ri.goff, ri.pairs, w.o_part, w.l_part, w.status, st);
+        rc = ret_fwd_tc(d, Q, Kp, Vp, off_k, ri.goff, ri.pairs, bsel, w.o_part, w.l_part, w.status, st);
         if (rc != MUSE_OK) return rc;
       } else {
         MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fl_smem));
@@ -599,23 +626,26 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
   prof_mark("k_merge", st);
   if (kTensor)
     k_merge<T, D, __nv_bfloat16><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.o_far, w.lse_far, w.o_loc, w.lse_loc,
-                                                                       (const __nv_bfloat16*)w.o_part, w.l_part, sel, O, LSE);
+                                                                       (const __nv_bfloat16*)w.o_part, w.l_part, two_level ? w.o_near : nullptr,
+                                                                       two_level ? w.lse_near : nullptr, sel, O, LSE);
   else
-    k_merge<T, D, float><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.o_far, w.lse_far, w.o_loc, w.lse_loc, w.o_part, w.l_part, sel, O, LSE);
+    k_merge<T, D, float><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.o_far, w.lse_far, w.o_loc, w.lse_loc, w.o_part, w.l_part, nullptr, nullptr,
+                                                               sel, O, LSE);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }
 
 int attn_fwd(const Dims& d, int dtype, const void* Q, const void* K, const void* V, const int32_t* assign_q,
              const float* qbar, const int32_t* off_k, const int32_t* perm_k, const void* summaries,
-             const int32_t* sel_in, void* O, float* LSE, int32_t* sel_out, void* ws, cudaStream_t st) {
+             const int32_t* sel_in, const int32_t* bsel_in, void* O, float* LSE, int32_t* sel_out, int32_t* bsel_out, void* ws,
+             cudaStream_t st) {
   typedef __nv_bfloat16 bf;
   if (dtype == MUSE_F32) {
-    if (d.D == 64) return attn_fwd_t<float, 64>(d, (const float*)Q, (const float*)K, (const float*)V, assign_q, qbar, off_k, perm_k, summaries, sel_in, (float*)O, LSE, sel_out, ws, dtype, st);
-    return attn_fwd_t<float, 128>(d, (const float*)Q, (const float*)K, (const float*)V, assign_q, qbar, off_k, perm_k, summaries, sel_in, (float*)O, LSE, sel_out, ws, dtype, st);
+    if (d.D == 64) return attn_fwd_t<float, 64>(d, (const float*)Q, (const float*)K, (const float*)V, assign_q, qbar, off_k, perm_k, summaries, sel_in, bsel_in, (float*)O, LSE, sel_out, bsel_out, ws, dtype, st);
+    return attn_fwd_t<float, 128>(d, (const float*)Q, (const float*)K, (const float*)V, assign_q, qbar, off_k, perm_k, summaries, sel_in, bsel_in, (float*)O, LSE, sel_out, bsel_out, ws, dtype, st);
   }
-  if (d.D == 64) return attn_fwd_t<bf, 64>(d, (const bf*)Q, (const bf*)K, (const bf*)V, assign_q, qbar, off_k, perm_k, summaries, sel_in, (bf*)O, LSE, sel_out, ws, dtype, st);
-  return attn_fwd_t<bf, 128>(d, (const bf*)Q, (const bf*)K, (const bf*)V, assign_q, qbar, off_k, perm_k, summaries, sel_in, (bf*)O, LSE, sel_out, ws, dtype, st);
+  if (d.D == 64) return attn_fwd_t<bf, 64>(d, (const bf*)Q, (const bf*)K, (const bf*)V, assign_q, qbar, off_k, perm_k, summaries, sel_in, bsel_in, (bf*)O, LSE, sel_out, bsel_out, ws, dtype, st);
+  return attn_fwd_t<bf, 128>(d, (const bf*)Q, (const bf*)K, (const bf*)V, assign_q, qbar, off_k, perm_k, summaries, sel_in, bsel_in, (bf*)O, LSE, sel_out, bsel_out, ws, dtype, st);
 }
 
 }  // namespace muse

@@ -23,6 +23,7 @@ struct Dims {
   int Bs;       // block size N / S
   int causal, sel_mode, agg_grad;
   int dipole;   // 1: untilted pre-merged dipole correction of the far field (needs m == 0)
+  int k2;       // spatial selection: 0 = every earlier block of a selected cluster is retrieved; > 0 = only the k2 best (causal only)
   float sigma;
   HeadMap hm;
 };
@@ -150,13 +151,19 @@ int dipole_apply(const Dims& d, int dtype, const void* Q, const float* qbar, con
 //   bf16 mode: kappa = khi + klo, two bf16 planes [D] (tensor-core operands that keep ~16 bits
 //              of mantissa, so discrete top-m decisions match fp64); nu one bf16 plane [D]
 //   cbar (dipole only): merged dipole matrices [B,Hq,SB,Cq][D value dims][D key dims], fp32 or bf16
-struct SummLayout { size_t mu, beta, khi, klo, nu, Kp, Vp, cbar, total; };
+//   blk (k2 > 0 only): a second set mu | beta | kappa (hi, lo) | nu with the same shapes holding the PER-BLOCK
+//              (pre-accumulation) summaries: plane s = the summary of the keys of block s alone
+struct SummLayout { size_t mu, beta, khi, klo, nu, Kp, Vp, cbar, blk, blk_beta, blk_khi, blk_klo, blk_nu, total; };
 SummLayout summ_layout(const Dims& d, int dtype);
 
 struct SummPtrs { float* mu; float* beta; void* khi; void* klo; void* nu; };
 inline SummPtrs summ_ptrs(const SummLayout& L, const void* base_) {
   char* b = (char*)base_;
   return SummPtrs{(float*)(b + L.mu), (float*)(b + L.beta), b + L.khi, b + L.klo, b + L.nu};
+}
+inline SummPtrs summ_ptrs_blk(const SummLayout& L, const void* base_) {      // the per-block set (k2 > 0)
+  char* b = (char*)base_;
+  return SummPtrs{(float*)(b + L.blk), (float*)(b + L.blk_beta), b + L.blk_khi, b + L.blk_klo, b + L.blk_nu};
 }
 // ST = storage element type of kappa / nu (float or bf16); idx = element index (entry * D + d), d % 4 == 0
 template <class ST> __device__ __forceinline__ float4 ld_kappa4(const SummPtrs& s, size_t idx);
@@ -185,8 +192,8 @@ template <class ST> __device__ __forceinline__ void st_nu4(const SummPtrs& s, si
 
 int attn_fwd(const Dims& d, int dtype, const void* Q, const void* K, const void* V,
              const int32_t* assign_q, const float* qbar, const int32_t* off_k, const int32_t* perm_k,
-             const void* summaries, const int32_t* sel_in, void* O, float* LSE, int32_t* sel_out,
-             void* ws, cudaStream_t st);
+             const void* summaries, const int32_t* sel_in, const int32_t* bsel_in, void* O, float* LSE, int32_t* sel_out,
+             int32_t* bsel_out, void* ws, cudaStream_t st);
 size_t attn_fwd_ws_bytes(const Dims& d, int dtype);
 
 int attn_bwd(const Dims& d, int dtype, const void* Q, const void* K, const void* V, const void* O,

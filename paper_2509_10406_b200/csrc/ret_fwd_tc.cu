@@ -64,7 +64,7 @@ template <int D>
 __global__ void __launch_bounds__(rf::kThreads, 2)
 k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, const bf16* __restrict__ Vp,
                    const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
-                   bf16* __restrict__ o_part, float* __restrict__ l_part, int* __restrict__ status) {
+                   const int32_t* __restrict__ bsel, bf16* __restrict__ o_part, float* __restrict__ l_part, int* __restrict__ status) {
   using namespace rf;
   typedef Smem<D> SM;
   constexpr int CPR = D / 8;                               // 16-byte chunks per row
@@ -166,7 +166,27 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
         int pid_n, last_n;
         tile_ids(tile + nsub, pid_n, last_n);
         const int nk = visible(last, kc), nk16 = (nk + 15) & ~15;      // the tile's last pair has the latest plane: it sees the most keys
-        const int vis = pid >= 0 ? visible(pid, kc) : 0;
+        // which of the sweep's 128 key columns this row sees: the cluster's keys of the earlier blocks (a prefix), or,
+        // with spatial block selection (k2 > 0), the buckets of the chosen blocks only (Section "Two-Level Retrieval")
+        uint32_t vm[4] = {0u, 0u, 0u, 0u};
+        auto set_range = [&](int lo, int hi) {               // columns [lo, hi) of the sweep
+          lo = max(lo, 0); hi = min(hi, kKeys);
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            const int a = max(lo - 32 * g, 0), z = min(hi - 32 * g, 32);
+            if (z > a) vm[g] |= (z - a >= 32 ? 0xffffffffu : ((1u << (z - a)) - 1u) << a);
+          }
+        };
+        if (pid >= 0) {
+          if (dm.k2 == 0) set_range(0, visible(pid, kc));
+          else {
+            const int bq = (pid / dm.m) / dm.Bs;             // the query's block: only earlier blocks count
+            for (int e = 0; e < dm.k2; ++e) {
+              const int bb = __ldg(bsel + (pbase + pid) * dm.k2 + e);
+              if (bb >= 0 && bb < bq) set_range(ok[bb] - k0 - kc, ok[bb + 1] - k0 - kc);
+            }
+          }
+        }
         const float lse_old = (!first && pid >= 0) ? l_part[pbase + pid] : -INFINITY;
         float M = -INFINITY, l = 0.f;
         RFCLK(1)
@@ -180,9 +200,9 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
           for (int g = 0; 32 * g < nk16; ++g) {
             float sv[32];
             tc::tmem_ld32(tl + SM::cS + 32 * g, sv);
-            const int vg = vis - 32 * g;
+            const uint32_t w = vm[g];
 #pragma unroll
-            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, i < vg ? sv[i] : -INFINITY);
+            for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (w >> i) & 1u ? sv[i] : -INFINITY);
           }
           M = mx * scale2;                                 // (scale2 > 0)
           const float base = M == -INFINITY ? 0.f : M;
@@ -190,12 +210,12 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
           for (int g = 0; 32 * g < nk16; ++g) {
             float sv[32];
             tc::tmem_ld32(tl + SM::cS + 32 * g, sv);
-            const int vg = vis - 32 * g;
+            const uint32_t w = vm[g];
             uint32_t pk2[16];
 #pragma unroll
             for (int i = 0; i < 32; i += 2) {
-              const float e0 = i < vg ? tc::fast_exp2(fmaf(sv[i], scale2, -base)) : 0.f;
-              const float e1 = i + 1 < vg ? tc::fast_exp2(fmaf(sv[i + 1], scale2, -base)) : 0.f;
+              const float e0 = (w >> i) & 1u ? tc::fast_exp2(fmaf(sv[i], scale2, -base)) : 0.f;
+              const float e1 = (w >> (i + 1)) & 1u ? tc::fast_exp2(fmaf(sv[i + 1], scale2, -base)) : 0.f;
               l += e0 + e1;
               __nv_bfloat162 b2 = __floats2bfloat162_rn(e0, e1);
               pk2[i / 2] = *reinterpret_cast<uint32_t*>(&b2);
@@ -359,16 +379,16 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
 }
 
 int ret_fwd_pairs_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
-                     const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st) {
+                     const int32_t* pairs, const int32_t* bsel, void* o_part, float* l_part, int* status, cudaStream_t st) {
   const dim3 grid(d.Ck, rf::kSplit, d.B * d.Hq);
   prof_mark("k_ret_fwd_pairs_tc", st);
   if (d.D == 128) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_pairs_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, rf::Smem<128>::total));
-    k_ret_fwd_pairs_tc<128><<<grid, rf::kThreads, rf::Smem<128>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs,
+    k_ret_fwd_pairs_tc<128><<<grid, rf::kThreads, rf::Smem<128>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs, bsel,
                                                                           (bf16*)o_part, l_part, status);
   } else {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_pairs_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, rf::Smem<64>::total));
-    k_ret_fwd_pairs_tc<64><<<grid, rf::kThreads, rf::Smem<64>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs,
+    k_ret_fwd_pairs_tc<64><<<grid, rf::kThreads, rf::Smem<64>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs, bsel,
                                                                         (bf16*)o_part, l_part, status);
   }
   MUSE_LAUNCH_OK();

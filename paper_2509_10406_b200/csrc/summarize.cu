@@ -8,7 +8,7 @@ namespace muse {
 
 bool summarize_tc_supported(const Dims& d, int dtype);
 int summarize_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const float* qbar, const SummPtrs& sp,
-                 void* qsplit, int* status, cudaStream_t stream);
+                 int per_block, void* qsplit, int* status, cudaStream_t stream);
 
 SummLayout summ_layout(const Dims& d, int dtype) {
   const size_t es = dtype == MUSE_F32 ? 4 : 2;
@@ -23,7 +23,16 @@ SummLayout summ_layout(const Dims& d, int dtype) {
   L.Kp = up(L.nu + ent * d.D * es);
   L.Vp = up(L.Kp + (size_t)d.B * d.Hkv * d.N * d.D * es);
   L.cbar = up(L.Vp + (size_t)d.B * d.Hkv * d.N * d.D * es);
-  L.total = up(L.cbar + (d.dipole ? (size_t)d.B * d.Hq * d.SB * d.Cq * d.D * d.D * es : 0));
+  L.blk = up(L.cbar + (d.dipole ? (size_t)d.B * d.Hq * d.SB * d.Cq * d.D * d.D * es : 0));
+  L.blk_beta = L.blk_khi = L.blk_klo = L.blk_nu = L.blk;
+  L.total = L.blk;
+  if (d.k2 > 0) {                                       // per-block summaries beside the accumulated ones
+    L.blk_beta = up(L.blk + ent * sizeof(float));
+    L.blk_khi = up(L.blk_beta + ent * sizeof(float));
+    L.blk_klo = up(L.blk_khi + ent * d.D * es);
+    L.blk_nu = dtype == MUSE_F32 ? L.blk_klo : up(L.blk_klo + ent * d.D * es);
+    L.total = up(L.blk_nu + ent * d.D * es);
+  }
   return L;
 }
 
@@ -78,7 +87,7 @@ constexpr int kSumI = 64, kSumKC = 16, kSumThreads = 256;
 template <class T, int D>
 __global__ void __launch_bounds__(kSumThreads)
 k_summarize(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const int32_t* __restrict__ off_k,
-            const float* __restrict__ qbar, SummPtrs sp) {
+            const float* __restrict__ qbar, SummPtrs sp, int per_block) {
   constexpr int LDQ = D + 4, LDKV = 2 * D + 4, LDL = kSumKC + 1, NV = 2 * D / 32;
   extern __shared__ float smf[];
   float* qb = smf;                         // [64][LDQ]  sigma * qbar tile
@@ -111,6 +120,16 @@ k_summarize(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const i
 
   for (int b = 0; b < dm.SB; ++b) {
     const int p0 = off[b], p1 = off[b + 1];
+    if (per_block) {                                    // the summary of block b alone: the running state starts afresh
+#pragma unroll
+      for (int a = 0; a < 2; ++a) {
+        M[a] = -INFINITY; s[a] = 0.f;
+#pragma unroll
+        for (int k = 0; k < NV; ++k)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) acc[a][k][c] = 0.f;
+      }
+    }
     for (int c0 = p0; c0 < p1; c0 += kSumKC) {
       const int n = min(kSumKC, p1 - c0);
       __syncthreads();
@@ -197,7 +216,7 @@ k_summarize(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const i
 
 template <class T, int D>
 static int summarize_planes(const Dims& d, int dtype, const T* Kp, const T* Vp, const int32_t* off_k, const float* qbar,
-                            const SummLayout& L, char* base, void* qsplit, int32_t* status, cudaStream_t st);
+                            const SummPtrs& sp, int per_block, void* qsplit, int32_t* status, cudaStream_t st);
 
 // assign_k == nullptr: off_k and perm_k are inputs (the keys are already bucketed: the backward pass
 // rebuilding the summaries it was not given); `status` then points at the caller's status words.
@@ -231,21 +250,22 @@ static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const i
   }
   if (d.SB == 0) return MUSE_OK;
   void* qsplit = ar.take<__nv_bfloat16>(2 * (size_t)d.B * d.Hq * d.Cq * d.D);   // split centroids for the tensor kernel
-  rc = summarize_planes<T, D>(d, dtype, Kp, Vp, off_k, qbar, L, base, qsplit, status, st);
+  rc = summarize_planes<T, D>(d, dtype, Kp, Vp, off_k, qbar, summ_ptrs(L, base), 0, qsplit, status, st);
+  if (rc == MUSE_OK && d.k2 > 0) rc = summarize_planes<T, D>(d, dtype, Kp, Vp, off_k, qbar, summ_ptrs_blk(L, base), 1, qsplit, status, st);
   if (rc != MUSE_OK || !d.dipole) return rc;
   return dipole_build(d, dtype, Kp, Vp, off_k, summ_ptrs(L, base).mu, base + L.cbar, (char*)ws + ar.used, status, st);
 }
 
 template <class T, int D>
 static int summarize_planes(const Dims& d, int dtype, const T* Kp, const T* Vp, const int32_t* off_k, const float* qbar,
-                            const SummLayout& L, char* base, void* qsplit, int32_t* status, cudaStream_t st) {
+                            const SummPtrs& sp, int per_block, void* qsplit, int32_t* status, cudaStream_t st) {
   if (summarize_tc_supported(d, dtype) && !path_forced(kForceSummFwdSimt))
-    return summarize_tc(d, Kp, Vp, off_k, qbar, summ_ptrs(L, base), qsplit, status, st);
+    return summarize_tc(d, Kp, Vp, off_k, qbar, sp, per_block, qsplit, status, st);
   const size_t smem = (size_t)(kSumI * (D + 4) + kSumKC * (2 * D + 4) + kSumI * (kSumKC + 1)) * sizeof(float);
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   dim3 grid(d.Ck, cdiv(d.Cq, kSumI), d.B * d.Hq);
   prof_mark("k_summarize", st);
-  k_summarize<T, D><<<grid, kSumThreads, smem, st>>>(d, Kp, Vp, off_k, qbar, summ_ptrs(L, base));
+  k_summarize<T, D><<<grid, kSumThreads, smem, st>>>(d, Kp, Vp, off_k, qbar, sp, per_block);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }

@@ -55,7 +55,8 @@ __global__ void __launch_bounds__(st::THREADS, 1)
 k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_constant__ CUtensorMap tm_V,
                const __grid_constant__ CUtensorMap tm_okhi, const __grid_constant__ CUtensorMap tm_oklo,
                const __grid_constant__ CUtensorMap tm_onu, const __grid_constant__ CUtensorMap tm_qhi,
-               const __grid_constant__ CUtensorMap tm_qlo, const int32_t* __restrict__ off_k, SummPtrs sp, int* __restrict__ status) {
+               const __grid_constant__ CUtensorMap tm_qlo, const int32_t* __restrict__ off_k, SummPtrs sp, int per_block,
+               int* __restrict__ status) {
   using namespace st;
   typedef Lay<D> LY;
   constexpr int G = LY::G, HD = D / 2, kTile = LY::kTile;
@@ -122,6 +123,11 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
   if (tid == 32) issue_after(off[0]);
   for (int pl = 0; pl < dm.SB && ok; ++pl) {
     const int p0 = off[pl], p1 = off[pl + 1];
+    if (per_block) {                                     // the summary of block pl alone: the running state starts afresh
+      M = -INFINITY; s = 0.f; T = 0.f;
+#pragma unroll
+      for (int d = 0; d < D; ++d) acc[d] = 0.f;
+    }
     for (int c0 = p0; c0 < p1 && ok; c0 += NU) {
       const int nk = min(NU, p1 - c0);
       PCLK(0)
@@ -272,7 +278,7 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
 bool summarize_tc_supported(const Dims& d, int dtype) { return dtype == MUSE_BF16 && (d.D == 64 || d.D == 128); }
 
 int summarize_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const float* qbar, const SummPtrs& sp,
-                 void* qsplit, int* status, cudaStream_t stream) {
+                 int per_block, void* qsplit, int* status, cudaStream_t stream) {
   // qsplit: 2 * B*Hq*Cq*D bf16 of scratch for the split centroids
   bf16* qhi = (bf16*)qsplit;
   bf16* qlo = qhi + (size_t)d.B * d.Hq * d.Cq * d.D;
@@ -298,10 +304,10 @@ int summarize_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* o
   const dim3 grid(d.Ck, cdiv(d.Cq, st::TI), d.B * d.Hq);
   if (d.D == 128) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, st::Lay<128>::total));
-    k_summarize_tc<128><<<grid, st::THREADS, st::Lay<128>::total, stream>>>(d, tK, tV, okhi, oklo, onu, tqh, tql, off_k, sp, status);
+    k_summarize_tc<128><<<grid, st::THREADS, st::Lay<128>::total, stream>>>(d, tK, tV, okhi, oklo, onu, tqh, tql, off_k, sp, per_block, status);
   } else {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_summarize_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, st::Lay<64>::total));
-    k_summarize_tc<64><<<grid, st::THREADS, st::Lay<64>::total, stream>>>(d, tK, tV, okhi, oklo, onu, tqh, tql, off_k, sp, status);
+    k_summarize_tc<64><<<grid, st::THREADS, st::Lay<64>::total, stream>>>(d, tK, tV, okhi, oklo, onu, tqh, tql, off_k, sp, per_block, status);
   }
   MUSE_LAUNCH_OK();
   return MUSE_OK;

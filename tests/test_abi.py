@@ -38,12 +38,15 @@ def test_workspace_sizes_and_layout(mb):
     assert sizes[4] >= ent * (3 * 128 * 2 + 8) + 2 * 16 * 65536 * 128 * 2
     off = mb.muse_summaries_layout(p)
     assert off[0] == 0 and off[1] >= ent * 4 and off[3] - off[2] >= ent * 128 * 2 and all(o % 256 == 0 for o in off)
-    assert len(off) == 8 and list(off) == sorted(off)
+    assert len(off) == 9 and list(off) == sorted(off) and off[8] == sizes[4]        # no per-block set without k2
+    p2 = mb.make_params(B=1, Hq=16, Hkv=16, N=65536, D=128, Cq=256, Ck=1024, m=32, k2=1)
+    off2 = mb.muse_summaries_layout(p2)
+    assert mb.muse_workspace_bytes(p2)[4] - off2[8] >= ent * (3 * 128 * 2 + 8)      # the per-block set has the same size
     assert all(s % 256 == 0 for s in sizes)
 
 
 @pytest.mark.parametrize("kw,code", [
-    (dict(D=96), -2), (dict(m=2000), -1), (dict(N=1001), -1), (dict(Cq=0), -1), (dict(k2=1), -2),
+    (dict(D=96), -2), (dict(m=2000), -1), (dict(N=1001), -1), (dict(Cq=0), -1), (dict(k2=9), -2), (dict(k2=1, dtype="f32"), -2),
     (dict(dipole=1), -2), (dict(dipole=2), -1), (dict(Hq=3, Hkv=2), -1), (dict(m=65, Ck=128), -2), (dict(Ck=8192, N=16384), -2),
 ])
 def test_invalid_parameters_are_rejected_on_the_host(mb, kw, code):
@@ -64,7 +67,7 @@ def test_null_and_small_workspace_are_rejected(mb):
     assert L.muse_summarize(ctypes.byref(p), fake, fake, fake, fake, fake, fake, z, z, z, fake, fake, 16, z) == -3
     # the three untilted outputs come together
     assert L.muse_summarize(ctypes.byref(p), fake, fake, fake, fake, fake, fake, fake, z, z, fake, fake, 1 << 30, z) == -1
-    assert L.muse_attn_fwd(ctypes.byref(p), fake, fake, fake, fake, fake, fake, fake, fake, z, fake, fake, z, fake, 16, z) == -3
+    assert L.muse_attn_fwd(ctypes.byref(p), fake, fake, fake, fake, fake, fake, fake, fake, z, z, fake, fake, z, z, fake, 16, z) == -3
     odd = ctypes.c_void_p(4100)
     assert L.muse_summarize(ctypes.byref(p), odd, fake, fake, fake, fake, fake, z, z, z, fake, fake, 1 << 30, z) == -1
     # backward without summaries needs the larger scratch

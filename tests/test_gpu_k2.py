@@ -1,0 +1,115 @@
+"""GPU parity of the two-level retrieval (Section "Two-Level Retrieval": inside every selected cluster only the
+k2 best-scoring earlier blocks are retrieved exactly, the others enter through their per-block summaries; Section
+"Output merging": the four-way merge) against the fp64 oracle, forward pass, bf16 mode (2e-2 relative max-abs),
+with cluster and block selections forced both ways."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import muse_oracle as orc
+from tests.gpu_util import Case, to_dev, to_np, tol, rel_err, kernels_launched
+from tests.test_gpu_cluster import CASES
+from tests.test_gpu_forward import TC
+
+pytestmark = pytest.mark.gpu
+
+K2_CASES = {"d128": CASES["d128"], "tc": TC["tc"], "tc_d64": TC["tc_d64"]}
+
+
+def _run(mb, c, p, buf, Q, K, V, qbar32, sel_in=None, bsel_in=None):
+    mb.muse_attn_fwd(p, Q, K, V, to_dev(c.a_q, "i"), to_dev(qbar32, "f32"), buf.off_k, buf.perm_k, buf.summaries,
+                     None if sel_in is None else to_dev(sel_in, "i"), buf.O, buf.LSE, buf.sel, buf.ws,
+                     bsel_in=None if bsel_in is None else to_dev(bsel_in, "i"), bsel_out=buf.bsel)
+    torch.cuda.synchronize()
+    assert mb.muse_status(buf.ws) == 0
+    return to_np(buf.O), to_np(buf.LSE), to_np(buf.sel)[..., :c.w.m], to_np(buf.bsel)
+
+
+@pytest.mark.parametrize("name", list(K2_CASES))
+@pytest.mark.parametrize("k2", [1, 2])
+def test_two_level_forward_matches_oracle(name, k2):
+    from paper_2509_10406_b200 import binding as mb
+    w = K2_CASES[name]
+    c = Case(w, gain=128.0)
+    qbar32 = c.qbar.astype(np.float32)
+    p = c.params(k2=k2)
+    buf = mb.MuseBuffers(p, backward=False)
+    Q, K, V, _ = c.dev()
+    with kernels_launched() as rec:
+        mb.muse_summarize(p, K, V, to_dev(c.a_k, "i"), to_dev(qbar32, "f32"), buf.off_k, buf.perm_k, buf.summaries, buf.ws)
+        O_free, L_free, sel_gpu, bsel_gpu = _run(mb, c, p, buf, Q, K, V, qbar32)
+    assert {"k_block_select", "k_ret_fwd_pairs_tc"} <= rec.names, sorted(rec.names)
+    t = tol(w.dtype)
+    kw = dict(sigma=c.sigma, S=w.S, Ck=w.Ck, m=w.m, k2=k2)
+    sel_orc = np.full((w.B, w.Hq, w.N, w.m), -1, np.int32)
+    bsel_orc = np.full((w.B, w.Hq, w.N, w.m, k2), -1, np.int32)
+    worst = dict(forced_gpu=0.0, forced_orc=0.0, block_rows_differ=0, pairs=0)
+    for b in range(w.B):
+        for h in range(w.Hq):
+            g = c.hm[h]
+            args = (c.Q[b, h], c.K[b, g], c.V[b, g], c.a_q[b, h], c.a_k[b, g], qbar32[b, h].astype(np.float64))
+            f = orc.forward(*args, **kw)
+            sel_orc[b, h], bsel_orc[b, h] = f["sel"], f["bsel"]
+            # the oracle forced to the GPU's cluster AND block selections
+            ff = orc.forward(*args, sel=sel_gpu[b, h], bsel=bsel_gpu[b, h], summ=f["summ"], **kw)
+            e = max(rel_err(O_free[b, h], ff["O"]), float(np.abs(L_free[b, h] - ff["LSE"]).max() / max(1.0, np.abs(ff["LSE"]).max())))
+            worst["forced_gpu"] = max(worst["forced_gpu"], e)
+            # the GPU's blocks are valid: earlier than the query's block, distinct, inside non-empty buckets of the cluster
+            Bs = w.N // w.S
+            cnt = np.zeros((w.Ck, w.S), np.int64)
+            np.add.at(cnt, (c.a_k[b, g], np.arange(w.N) // Bs), 1)
+            for tq in range(0, w.N, 37):
+                for k in range(w.m):
+                    j = sel_gpu[b, h, tq, k]
+                    bl = bsel_gpu[b, h, tq, k]; bl = bl[bl >= 0]
+                    assert j >= 0 or bl.size == 0
+                    assert len(set(bl.tolist())) == bl.size and np.all(bl < tq // Bs)
+                    if j >= 0:
+                        assert np.all(cnt[j, bl] > 0)
+                        assert bl.size == min(k2, int((cnt[j, :tq // Bs] > 0).sum()))
+            # free selections compared where the cluster selections agree slot for slot after sorting by cluster
+            for tq in range(0, w.N, 11):
+                so, sg = f["sel"][tq], sel_gpu[b, h, tq]
+                if set(so.tolist()) != set(sg.tolist()):
+                    continue
+                for k in range(w.m):
+                    if so[k] < 0:
+                        continue
+                    kg = int(np.nonzero(sg == so[k])[0][0])
+                    worst["pairs"] += 1
+                    worst["block_rows_differ"] += int(set(f["bsel"][tq, k].tolist()) != set(bsel_gpu[b, h, tq, kg].tolist()))
+    assert worst["forced_gpu"] <= t, worst
+    # the GPU forced to the oracle's cluster and block selections
+    O_f, _, _, _ = _run(mb, c, p, buf, Q, K, V, qbar32, sel_in=sel_orc, bsel_in=bsel_orc)
+    for b in range(w.B):
+        for h in range(w.Hq):
+            g = c.hm[h]
+            f = orc.forward(c.Q[b, h], c.K[b, g], c.V[b, g], c.a_q[b, h], c.a_k[b, g], qbar32[b, h].astype(np.float64),
+                            sel=sel_orc[b, h], bsel=bsel_orc[b, h], **kw)
+            worst["forced_orc"] = max(worst["forced_orc"], rel_err(O_f[b, h], f["O"]))
+    print(name, k2, worst)
+    assert worst["forced_orc"] <= t, worst
+    # block choices may differ from the oracle's only at near-ties of the block logits: a small fraction
+    assert worst["block_rows_differ"] <= 0.02 * worst["pairs"] + 2, worst
+
+
+def test_retrieving_every_block_equals_single_level():
+    """k2 >= S - 1 retrieves every earlier block of the selected clusters: the near field is empty and the result is
+    that of k2 = 0 (up to the order of the floating-point sums)."""
+    from paper_2509_10406_b200 import binding as mb
+    w = TC["tc"]
+    c = Case(w, gain=128.0)
+    qbar32 = c.qbar.astype(np.float32)
+    Q, K, V, _ = c.dev()
+    outs = []
+    for k2 in (0, w.S - 1):
+        p = c.params(k2=k2)
+        buf = mb.MuseBuffers(p, backward=False)
+        mb.muse_summarize(p, K, V, to_dev(c.a_k, "i"), to_dev(qbar32, "f32"), buf.off_k, buf.perm_k, buf.summaries, buf.ws)
+        mb.muse_attn_fwd(p, Q, K, V, to_dev(c.a_q, "i"), to_dev(qbar32, "f32"), buf.off_k, buf.perm_k, buf.summaries, None,
+                         buf.O, buf.LSE, buf.sel, buf.ws, bsel_out=buf.bsel)
+        torch.cuda.synchronize()
+        assert mb.muse_status(buf.ws) == 0
+        outs.append((to_np(buf.O), to_np(buf.LSE)))
+    assert rel_err(outs[1][0], outs[0][0]) <= 1e-2
+    assert np.abs(outs[1][1] - outs[0][1]).max() <= 1e-3 * max(1.0, np.abs(outs[0][1]).max())
