@@ -294,6 +294,8 @@ def main():
                     help="run the KV-head groups in this many sequential stages over one set of buffers "
                          "(0 = as few as keep the summaries under 64 GB)")
     ap.add_argument("--forward-only", action="store_true", help="time cluster + summarize + forward only")
+    ap.add_argument("--k2", type=int, default=0,
+                    help="spatial blocks retrieved inside each selected cluster (0 = all; > 0 is forward only)")
     ap.add_argument("--dipole", action="store_true",
                     help="far field with the dipole correction instead of retrieval (sets m = 0, forward only)")
     ap.add_argument("--ref-rows", type=int, default=128, help="sampled queries for the oracle timing")
@@ -309,6 +311,8 @@ def main():
         w = w.with_(m=args.m)
     if args.dipole:
         w = w.with_(m=0)
+        args.forward_only = True
+    if args.k2 > 0:
         args.forward_only = True
     if args.kmeans_iters is not None:
         w = w.with_(T=args.kmeans_iters)
@@ -351,7 +355,7 @@ def main():
         raise SystemExit("head staging needs B == 1 and a group count that divides the KV heads")
     hq, hkv = w.Hq // groups, w.Hkv // groups
     p = mb.make_params(B=w.B, Hq=hq, Hkv=hkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=w.m, n_blocks=w.S,
-                       dtype=w.dtype, kmeans_iters=w.T, dipole=int(args.dipole))
+                       dtype=w.dtype, kmeans_iters=w.T, dipole=int(args.dipole), k2=args.k2)
     buf = mb.MuseBuffers(p, backward=not args.forward_only)
     O_all = torch.empty_like(Q)
     dQ_all, dK_all, dV_all = (None, None, None) if args.forward_only else (torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V))
@@ -371,7 +375,7 @@ def main():
             mb.muse_summarize(p, Kg, Vg, buf.assign_k, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
             m_("summarize")
             mb.muse_attn_fwd(p, Qg, Kg, Vg, buf.assign_q, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, None,
-                             O_all[:, qs], buf.LSE, buf.sel, buf.ws)
+                             O_all[:, qs], buf.LSE, buf.sel, buf.ws, bsel_out=buf.bsel)
             m_("forward")
             if not args.forward_only:
                 mb.muse_attn_bwd(p, Qg, Kg, Vg, O_all[:, qs], buf.LSE, dO[:, qs], buf.assign_q, buf.qbar, buf.off_k,
@@ -451,7 +455,7 @@ def main():
             ep, ebuf = p, buf
         else:
             ep = mb.make_params(B=w.B, Hq=ehq, Hkv=ehkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=w.m, n_blocks=w.S,
-                                dtype=w.dtype, kmeans_iters=w.T, dipole=int(args.dipole))
+                                dtype=w.dtype, kmeans_iters=w.T, dipole=int(args.dipole), k2=args.k2)
             ebuf = mb.MuseBuffers(ep, backward=not args.forward_only)
         s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
 
@@ -479,7 +483,7 @@ def main():
                 cur.wait_event(e_v)
                 mb.muse_summarize(ep, Kg, Vg, ebuf.assign_k, ebuf.qbar, ebuf.off_k, ebuf.perm_k, ebuf.summaries, ebuf.ws)
                 mb.muse_attn_fwd(ep, Qg, Kg, Vg, ebuf.assign_q, ebuf.qbar, ebuf.off_k, ebuf.perm_k, ebuf.summaries, None,
-                                 O_all[:, qs], ebuf.LSE, ebuf.sel, ebuf.ws)
+                                 O_all[:, qs], ebuf.LSE, ebuf.sel, ebuf.ws, bsel_out=ebuf.bsel)
                 e_o = torch.cuda.Event(); e_o.record(cur)
                 with torch.cuda.stream(s_out):
                     s_out.wait_event(e_o)
@@ -568,8 +572,9 @@ def main():
 
             def dense():
                 o = F.scaled_dot_product_attention(q, k, v, is_causal=True)
-                o.backward(dO)
-                q.grad = k.grad = v.grad = None
+                if not args.forward_only:
+                    o.backward(dO)
+                    q.grad = k.grad = v.grad = None
                 return o
             dense(); torch.cuda.synchronize()
             ev0.record()
@@ -577,7 +582,7 @@ def main():
                 o_dense = dense()
             ev1.record(); torch.cuda.synchronize()
             dms = ev0.elapsed_time(ev1) / 3
-            context["dense_sdpa_fwd_bwd_ms"] = dms
+            context["dense_sdpa_forward_only_ms" if args.forward_only else "dense_sdpa_fwd_bwd_ms"] = dms
             context["speedup_vs_dense_sdpa"] = dms / ms
             if groups == 1 and O_first is not None:
                 # relative squared error of the approximation against exact attention, averaged over queries
@@ -639,7 +644,7 @@ def main():
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype,
             "data": "synthetic",
             "config": dict(workload_config(w, args.gain), head_stages=groups,
-                           dipole=int(args.dipole), passes="cluster+summarize+forward" if args.forward_only else "cluster+summarize+forward+backward"),
+                           dipole=int(args.dipole), k2=args.k2, passes="cluster+summarize+forward" if args.forward_only else "cluster+summarize+forward+backward"),
             "ms_per_step_median": statistics.median(per_step), "ms_per_step_best": min(per_step), "stages_ms": stages,
             "clocks": clocks, "e2e": e2e,
             "gpu_launches": launches, "roofline": roof, "cpu_baseline": cpu, "kernels": kernels, "context": context,

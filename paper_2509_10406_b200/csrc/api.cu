@@ -51,6 +51,7 @@ int resolve(const muse_params_t* p, Dims* d) {
   d->k2 = p->causal ? p->k2 : 0;                          // spatial selection needs spatial blocks
   if (d->k2 > 0 && S - 1 > 32) return MUSE_ERR_UNSUPPORTED;
   if (d->k2 > 0 && p->dtype != MUSE_BF16) return MUSE_ERR_UNSUPPORTED;   // built on the bf16 retrieval kernel
+  if (d->k2 > 0 && p->m * d->k2 > kMaxM) return MUSE_ERR_UNSUPPORTED;    // at most 64 retrieved buckets per query
   d->sigma = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->D);
   for (int h = 0; h < kMaxHeads; ++h) d->hm.g[h] = 0;
   for (int h = 0; h < p->Hq; ++h) {

@@ -724,7 +724,7 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
     if (rc != MUSE_OK) return rc;
     if (d.m > 0) {
       RetIndex ri;
-      rc = build_ret_index(d, sel, w.ret_scratch, &ri, st);
+      rc = build_ret_index(d, sel, nullptr, w.ret_scratch, &ri, st);
       if (rc != MUSE_OK) return rc;
       if (kTensor) {
         rc = ret_bwd_tc(d, Q, dO, Kp, Vp, LSE, w.delta, off_k, ri.goff, ri.pairs, w.dq_part, w.dK_perm, w.dV_perm, w.status, st);

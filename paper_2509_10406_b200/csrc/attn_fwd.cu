@@ -14,9 +14,9 @@ bool far_fwd_tc_supported(const Dims& d, int dtype);
 int far_fwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const int32_t* off_q, const int32_t* perm_q,
                const int32_t* sel_in, int32_t* sel_out, float* o_far, float* lse_far, int* status, cudaStream_t st);
 int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
-               const int32_t* pairs, const int32_t* bsel, void* o_part, float* l_part, int* status, cudaStream_t st);
-int block_select(const Dims& d, int dtype, const void* Q, const int32_t* assign_q, const int32_t* sel, const SummPtrs& sp,
-                 const int32_t* bsel_in, int32_t* bsel_out, float* o_near, float* lse_near, cudaStream_t st);
+               const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st);
+int block_select(const Dims& d, int dtype, const void* Q, const int32_t* assign_q, const int32_t* perm_q, const int32_t* sel,
+                 const SummPtrs& sp, const int32_t* bsel_in, int32_t* bsel_out, float* o_near, float* lse_near, cudaStream_t st);
 
 // plane of a query = index of the accumulated-summary plane it reads: block - 1 when causal
 // (block 0 sees no far field), 0 when non-causal.
@@ -30,47 +30,61 @@ __device__ __forceinline__ int query_plane(const Dims& d, int t) { return d.caus
 // Thread e handles (slot = e / N, query = e % N): the lanes of a warp are consecutive queries,
 // which often retrieve the same cluster in the same slot, so equal keys are combined with a warp
 // match and only one atomic per distinct key and warp reaches memory.
-__global__ void k_ret_count(Dims d, const int32_t* __restrict__ sel, int32_t* __restrict__ cnt) {
-  const int pq = blockIdx.y;
-  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  int key = -1;
-  if (e < (long long)d.N * d.m) {
-    const int t = (int)(e % d.N), k = (int)(e / d.N);
-    const int c = sel[((size_t)pq * d.N + t) * d.m + k];
-    const int pl = query_plane(d, t);
-    if (c >= 0 && c < d.Ck && pl >= 0) key = c * d.SB + pl;      // entries outside [0, Ck) count as "none"
-  }
-  const unsigned peers = __match_any_sync(0xffffffffu, key);
-  const int lane = threadIdx.x & 31;
-  if (key >= 0 && lane == __ffs(peers) - 1) atomicAdd(&cnt[(size_t)pq * d.SB * d.Ck + key], __popc(peers));
+// With spatial block selection (bsel != nullptr, k2 > 0) a pair is (query, slot, chosen block e2), its group the
+// BUCKET (cluster, chosen block) and its id (query * m + slot) * k2 + e2: the retrieval kernel then keeps one bucket
+// resident and every pair of the group sees all of it.
+__device__ __forceinline__ void ret_pair_key(const Dims& d, const int32_t* sel, const int32_t* bsel, int pq, long long e, int e2,
+                                             int& key, int& pid) {
+  key = -1; pid = 0;
+  if (e >= (long long)d.N * d.m) return;
+  const int t = (int)(e % d.N), k = (int)(e / d.N);
+  const size_t slot = ((size_t)pq * d.N + t) * d.m + k;
+  const int c = sel[slot];
+  const int pl = query_plane(d, t);
+  if (c < 0 || c >= d.Ck || pl < 0) return;                // entries outside [0, Ck) count as "none"
+  if (bsel == nullptr) { key = c * d.SB + pl; pid = t * d.m + k; return; }
+  const int bb = bsel[slot * d.k2 + e2];
+  if (bb < 0 || bb > pl) return;                           // (block bb is earlier than the query's block pl + 1)
+  key = c * d.SB + bb; pid = (t * d.m + k) * d.k2 + e2;
 }
 
-__global__ void k_ret_fill(Dims d, const int32_t* __restrict__ sel, int32_t* __restrict__ cursor,
+__global__ void k_ret_count(Dims d, const int32_t* __restrict__ sel, const int32_t* __restrict__ bsel, int32_t* __restrict__ cnt) {
+  const int pq = blockIdx.y;
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  const int lane = threadIdx.x & 31;
+  for (int e2 = 0; e2 < (bsel ? d.k2 : 1); ++e2) {
+    int key, pid;
+    ret_pair_key(d, sel, bsel, pq, e, e2, key, pid);
+    const unsigned peers = __match_any_sync(0xffffffffu, key);
+    if (key >= 0 && lane == __ffs(peers) - 1) atomicAdd(&cnt[(size_t)pq * d.SB * d.Ck + key], __popc(peers));
+  }
+}
+
+__global__ void k_ret_fill(Dims d, const int32_t* __restrict__ sel, const int32_t* __restrict__ bsel, int32_t* __restrict__ cursor,
                            int32_t* __restrict__ pairs) {
   const int pq = blockIdx.y;
   const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-  int key = -1, pid = 0;
-  if (e < (long long)d.N * d.m) {
-    const int t = (int)(e % d.N), k = (int)(e / d.N);
-    const int c = sel[((size_t)pq * d.N + t) * d.m + k];
-    const int pl = query_plane(d, t);
-    if (c >= 0 && c < d.Ck && pl >= 0) { key = c * d.SB + pl; pid = t * d.m + k; }
+  const int lane = threadIdx.x & 31;
+  const size_t npairs = (size_t)d.N * d.m * (bsel ? d.k2 : 1);
+  for (int e2 = 0; e2 < (bsel ? d.k2 : 1); ++e2) {
+    int key, pid;
+    ret_pair_key(d, sel, bsel, pq, e, e2, key, pid);
+    const unsigned peers = __match_any_sync(0xffffffffu, key);
+    const int leader = __ffs(peers) - 1;
+    int base = 0;
+    if (key >= 0 && lane == leader) base = atomicAdd(&cursor[(size_t)pq * d.SB * d.Ck + key], __popc(peers));
+    base = __shfl_sync(0xffffffffu, base, leader);
+    if (key >= 0) pairs[(size_t)pq * npairs + base + __popc(peers & ((1u << lane) - 1u))] = pid;
   }
-  const unsigned peers = __match_any_sync(0xffffffffu, key);
-  const int lane = threadIdx.x & 31, leader = __ffs(peers) - 1;
-  int base = 0;
-  if (key >= 0 && lane == leader) base = atomicAdd(&cursor[(size_t)pq * d.SB * d.Ck + key], __popc(peers));
-  base = __shfl_sync(0xffffffffu, base, leader);
-  if (key >= 0) pairs[(size_t)pq * d.N * d.m + base + __popc(peers & ((1u << lane) - 1u))] = pid;
 }
 
 size_t ret_index_elems(const Dims& d) {
-  // cursor [SB*Ck] + goff [SB*Ck+1] + pairs [N*m], each rounded up to 64 ints
+  // cursor [SB*Ck] + goff [SB*Ck+1] + pairs [N*m*max(k2,1)], each rounded up to 64 ints
   auto up = [](size_t x) { return (x + 63) & ~size_t(63); };
-  return up((size_t)d.SB * d.Ck) + up((size_t)d.SB * d.Ck + 1) + up((size_t)d.N * d.m);
+  return up((size_t)d.SB * d.Ck) + up((size_t)d.SB * d.Ck + 1) + up((size_t)d.N * d.m * (d.k2 > 0 ? d.k2 : 1));
 }
 
-int build_ret_index(const Dims& d, const int32_t* sel, int32_t* scratch, RetIndex* out, cudaStream_t st) {
+int build_ret_index(const Dims& d, const int32_t* sel, const int32_t* bsel, int32_t* scratch, RetIndex* out, cudaStream_t st) {
   auto up = [](size_t x) { return (x + 63) & ~size_t(63); };
   const int pq = d.B * d.Hq, nkeys = d.SB * d.Ck;
   out->cursor = scratch;
@@ -83,12 +97,12 @@ int build_ret_index(const Dims& d, const int32_t* sel, int32_t* scratch, RetInde
   MUSE_CUDA_OK(cudaMemsetAsync(out->cursor, 0, (size_t)pq * nkeys * sizeof(int32_t), st));
   dim3 grid(cdiv((long long)d.N * d.m > 0 ? d.N * d.m : 1, 256), pq);
   prof_mark("k_ret_count", st);
-  k_ret_count<<<grid, 256, 0, st>>>(d, sel, out->cursor);
+  k_ret_count<<<grid, 256, 0, st>>>(d, sel, bsel, out->cursor);
   MUSE_LAUNCH_OK();
   int rc = launch_scan(out->cursor, pq, nkeys, 1, out->goff, st);
   if (rc != MUSE_OK) return rc;
   prof_mark("k_ret_fill", st);
-  k_ret_fill<<<grid, 256, 0, st>>>(d, sel, out->cursor, out->pairs);
+  k_ret_fill<<<grid, 256, 0, st>>>(d, sel, bsel, out->cursor, out->pairs);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }
@@ -446,7 +460,7 @@ __global__ void k_merge(Dims dm, const float* __restrict__ o_far, const float* _
                         const float* __restrict__ o_loc, const float* __restrict__ lse_loc,
                         const PT* __restrict__ o_part, const float* __restrict__ l_part,
                         const float* __restrict__ o_near, const float* __restrict__ lse_near,
-                        const int32_t* __restrict__ sel, T* __restrict__ O, float* __restrict__ LSE) {
+                        const int32_t* __restrict__ sel, const int32_t* __restrict__ bsel, T* __restrict__ O, float* __restrict__ LSE) {
   const int pq = blockIdx.y;
   const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (t >= dm.N) return;
@@ -458,13 +472,14 @@ __global__ void k_merge(Dims dm, const float* __restrict__ o_far, const float* _
   // near field (component 2 of the merge): non-retrieved earlier blocks of the selected clusters; empty unless k2 > 0
   const float ln = (far_ok && lse_near != nullptr) ? lse_near[row] : -INFINITY;
   float mx = fmaxf(fmaxf(lf, ll), ln);
-  const int m = dm.m;
-  float lp_mine[2] = {-INFINITY, -INFINITY};        // slots lane, lane + 32
+  // retrieved partial results of this query: one per slot, or one per (slot, chosen block) with spatial block selection
+  const int kk = bsel != nullptr ? dm.k2 : 1, m = dm.m * kk;
+  float lp_mine[2] = {-INFINITY, -INFINITY};        // partials lane, lane + 32
   if (far_ok) {
 #pragma unroll
     for (int a = 0; a < 2; ++a) {
       const int s = lane + 32 * a;
-      if (s < m && sel[row * m + s] >= 0) lp_mine[a] = l_part[row * m + s];
+      if (s < m && sel[row * dm.m + s / kk] >= 0 && (bsel == nullptr || bsel[row * m + s] >= 0)) lp_mine[a] = l_part[row * m + s];
       mx = fmaxf(mx, lp_mine[a]);
     }
   }
@@ -544,8 +559,9 @@ static FwdWs fwd_ws(const Dims& d, Arena& ar) {
   w.lse_far = ar.take<float>(pq * d.N);
   w.o_loc = ar.take<float>(pq * d.N * d.D);
   w.lse_loc = ar.take<float>(pq * d.N);
-  w.o_part = ar.take<float>(pq * d.N * d.m * d.D);
-  w.l_part = ar.take<float>(pq * d.N * d.m);
+  const size_t mk = (size_t)d.m * (d.k2 > 0 ? d.k2 : 1);      // partial results per query
+  w.o_part = ar.take<float>(pq * d.N * mk * d.D);
+  w.l_part = ar.take<float>(pq * d.N * mk);
   const bool two_level = d.k2 > 0 && d.causal;
   w.bsel_tmp = ar.take<int32_t>(two_level ? pq * d.N * d.m * d.k2 : 0);
   w.o_near = ar.take<float>(two_level ? pq * d.N * d.D : 0);
@@ -605,15 +621,15 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
     }
     if (two_level) {
       // second level: the k2 best earlier blocks of every selected cluster, and the near field of the others
-      rc = block_select(d, dtype, Q, assign_q, sel, summ_ptrs_blk(L, base), bsel_in, bsel, w.o_near, w.lse_near, st);
+      rc = block_select(d, dtype, Q, assign_q, w.perm_q, sel, summ_ptrs_blk(L, base), bsel_in, bsel, w.o_near, w.lse_near, st);
       if (rc != MUSE_OK) return rc;
     }
     if (d.m > 0) {
       RetIndex ri;
-      rc = build_ret_index(d, sel, w.ret_scratch, &ri, st);
+      rc = build_ret_index(d, sel, bsel, w.ret_scratch, &ri, st);
       if (rc != MUSE_OK) return rc;
       if (kTensor) {
-        rc = ret_fwd_tc(d, Q, Kp, Vp, off_k, ri.goff, ri.pairs, bsel, w.o_part, w.l_part, w.status, st);
+        rc = ret_fwd_tc(d, Q, Kp, Vp, off_k, ri.goff, ri.pairs, w.o_part, w.l_part, w.status, st);
         if (rc != MUSE_OK) return rc;
       } else {
         MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fl_smem));
@@ -627,10 +643,10 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
   if (kTensor)
     k_merge<T, D, __nv_bfloat16><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.o_far, w.lse_far, w.o_loc, w.lse_loc,
                                                                        (const __nv_bfloat16*)w.o_part, w.l_part, two_level ? w.o_near : nullptr,
-                                                                       two_level ? w.lse_near : nullptr, sel, O, LSE);
+                                                                       two_level ? w.lse_near : nullptr, sel, bsel, O, LSE);
   else
     k_merge<T, D, float><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.o_far, w.lse_far, w.o_loc, w.lse_loc, w.o_part, w.l_part, nullptr, nullptr,
-                                                               sel, O, LSE);
+                                                               sel, nullptr, O, LSE);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }

@@ -436,14 +436,14 @@ int local_fwd_tc(const Dims& d, const void* Q, const void* K, const void* V, flo
 }
 
 int ret_fwd_pairs_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
-                     const int32_t* pairs, const int32_t* bsel, void* o_part, float* l_part, int* status, cudaStream_t st);
+                     const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st);
 
 int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
-               const int32_t* pairs, const int32_t* bsel, void* o_part, float* l_part, int* status, cudaStream_t st) {
+               const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st) {
   dim3 grid(d.Ck, d.SB * kRetFwdSplit, d.B * d.Hq);
   const int min_keys = 0;
   if (!path_forced(kForceRetFwdStream) || d.k2 > 0)           // (block selection exists in the pair kernel only)
-    return ret_fwd_pairs_tc(d, Q, Kp, Vp, off_k, goff, pairs, bsel, o_part, l_part, status, st);
+    return ret_fwd_pairs_tc(d, Q, Kp, Vp, off_k, goff, pairs, o_part, l_part, status, st);
   prof_mark("k_ret_fwd_tc", st);
   if (d.D == 128) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, FwdTcSmem<128>::total));

@@ -206,6 +206,7 @@ size_t attn_bwd_ws_bytes(const Dims& d, int dtype);
 // (query block - 1, key cluster).  pair id = t * m + slot.
 struct RetIndex { int32_t* goff; int32_t* pairs; int32_t* cursor; };
 size_t ret_index_elems(const Dims& d);     // int32 elements per query head
-int build_ret_index(const Dims& d, const int32_t* sel, int32_t* scratch, RetIndex* out, cudaStream_t st);
+// bsel != nullptr (k2 > 0): groups are the (cluster, chosen block) buckets, pair id = (t * m + slot) * k2 + e
+int build_ret_index(const Dims& d, const int32_t* sel, const int32_t* bsel, int32_t* scratch, RetIndex* out, cudaStream_t st);
 
 }  // namespace muse

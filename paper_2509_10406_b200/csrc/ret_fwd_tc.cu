@@ -64,7 +64,7 @@ template <int D>
 __global__ void __launch_bounds__(rf::kThreads, 2)
 k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__ Kp, const bf16* __restrict__ Vp,
                    const int32_t* __restrict__ off_k, const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs,
-                   const int32_t* __restrict__ bsel, bf16* __restrict__ o_part, float* __restrict__ l_part, int* __restrict__ status) {
+                   bf16* __restrict__ o_part, float* __restrict__ l_part, int* __restrict__ status) {
   using namespace rf;
   typedef Smem<D> SM;
   constexpr int CPR = D / 8;                               // 16-byte chunks per row
@@ -74,16 +74,21 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   __shared__ int32_t ok_s[kOkCache];
   __shared__ int32_t tok_s[kPairs];                        // tokens of the tile being gathered
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int j = blockIdx.x, sub = blockIdx.y, pq = blockIdx.z;
+  // Without spatial block selection the CTA owns a key cluster and its pairs of every plane (a query sees the cluster's
+  // keys of the earlier blocks).  With it (k2 > 0) the CTA owns one BUCKET (cluster, block bb): its pairs are the
+  // (query, slot, chosen block) triples that chose this block, and every one of them sees the whole bucket.
+  const bool bucket = dm.k2 > 0;
+  const int j = bucket ? blockIdx.x / dm.SB : blockIdx.x, bb = bucket ? blockIdx.x % dm.SB : 0, sub = blockIdx.y, pq = blockIdx.z;
+  const int mk = dm.m * (bucket ? dm.k2 : 1);              // partial results per query
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int ngroups = dm.SB * dm.Ck;
-  const int32_t* go = goff + (size_t)pq * (ngroups + 1) + (size_t)j * dm.SB;   // the cluster's pairs: plane pl is [go[pl], go[pl + 1])
-  const int g0 = go[0], g1 = go[dm.SB];
+  const int32_t* go = goff + (size_t)pq * (ngroups + 1) + (size_t)j * dm.SB + bb;   // the group's pairs: plane pl is [go[pl], go[pl + 1])
+  const int g0 = go[0], g1 = go[bucket ? 1 : dm.SB];
   const int ntiles = (g1 - g0 + kPairs - 1) / kPairs;
   const int nsub = min(kSplit, max(1, ntiles / kTilesPerCta));           // tiles are dealt round-robin to nsub CTAs
   if (ntiles == 0 || sub >= nsub) return;
   const int32_t* okg = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;   // okg[b]: first key of bucket (j, b)
-  const int k0 = okg[0], kall = okg[dm.SB] - k0;                         // keys that some plane sees
+  const int k0 = okg[bb], kall = (bucket ? okg[bb + 1] : okg[dm.SB]) - k0;   // keys that some pair of the group sees
   const int32_t* ok = dm.S + 1 <= kOkCache ? ok_s : okg;
   if (dm.S + 1 <= kOkCache)
     for (int b = tid; b <= dm.S; b += kThreads) ok_s[b] = okg[b];
@@ -102,12 +107,13 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   const bf16* Qb = Q + (size_t)pq * dm.N * D;
   const bf16* Kb = Kp + ((size_t)pk * dm.N + k0) * D;
   const bf16* Vb = Vp + ((size_t)pk * dm.N + k0) * D;
-  const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
-  const size_t pbase = (size_t)pq * dm.N * dm.m;
+  const int32_t* pr = pairs + (size_t)pq * dm.N * mk;
+  const size_t pbase = (size_t)pq * dm.N * mk;
   bool ok_ = true;                                         // false once a bounded wait ran out (every role still walks all its tiles)
   auto wait = [&](uint64_t* bar, uint32_t parity) { if (ok_ && !tc::mbar_wait(bar, parity)) ok_ = false; };
   // keys of sweep `kc` that the query of pair `pid` sees (its block's prefix of the cluster)
   auto visible = [&](int pid, int kc) {
+    if (bucket) return min(kKeys, max(0, kall - kc));
     const int tok = pid / dm.m;
     return min(kKeys, max(0, ok[dm.causal ? tok / dm.Bs : 1] - k0 - kc));
   };
@@ -126,7 +132,7 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
     const bool first = kc == 0;
     // later sweeps pass over the tiles of planes that see none of the sweep's keys (a prefix of the cluster's tiles)
     int tile_lo = 0;
-    if (!first) {
+    if (!first && !bucket) {
       int pl = 0;
       while (pl + 1 < dm.SB && ok[pl + 1] - k0 <= kc) ++pl;
       tile_lo = (go[pl] - g0) / kPairs;
@@ -166,8 +172,7 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
         int pid_n, last_n;
         tile_ids(tile + nsub, pid_n, last_n);
         const int nk = visible(last, kc), nk16 = (nk + 15) & ~15;      // the tile's last pair has the latest plane: it sees the most keys
-        // which of the sweep's 128 key columns this row sees: the cluster's keys of the earlier blocks (a prefix), or,
-        // with spatial block selection (k2 > 0), the buckets of the chosen blocks only (Section "Two-Level Retrieval")
+        // which of the sweep's 128 key columns this row sees (a prefix: the cluster's keys of the earlier blocks, or the bucket)
         uint32_t vm[4] = {0u, 0u, 0u, 0u};
         auto set_range = [&](int lo, int hi) {               // columns [lo, hi) of the sweep
           lo = max(lo, 0); hi = min(hi, kKeys);
@@ -177,16 +182,7 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
             if (z > a) vm[g] |= (z - a >= 32 ? 0xffffffffu : ((1u << (z - a)) - 1u) << a);
           }
         };
-        if (pid >= 0) {
-          if (dm.k2 == 0) set_range(0, visible(pid, kc));
-          else {
-            const int bq = (pid / dm.m) / dm.Bs;             // the query's block: only earlier blocks count
-            for (int e = 0; e < dm.k2; ++e) {
-              const int bb = __ldg(bsel + (pbase + pid) * dm.k2 + e);
-              if (bb >= 0 && bb < bq) set_range(ok[bb] - k0 - kc, ok[bb + 1] - k0 - kc);
-            }
-          }
-        }
+        if (pid >= 0) set_range(0, visible(pid, kc));
         const float lse_old = (!first && pid >= 0) ? l_part[pbase + pid] : -INFINITY;
         float M = -INFINITY, l = 0.f;
         RFCLK(1)
@@ -346,7 +342,7 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
         if (nk > 0) {
           if (nproc > 0) wait(&bars.q_empty, (nproc - 1) & 1);   // the previous tile's first product has read the buffer
 #pragma unroll
-          for (int u = 0; u < RPT; ++u) tok_s[g + u * kGather] = pa[u] >= 0 ? pa[u] / dm.m : -1;
+          for (int u = 0; u < RPT; ++u) tok_s[g + u * kGather] = pa[u] >= 0 ? pa[u] / mk : -1;
           tc::named_bar_sync(1, kGather);
 #pragma unroll 4
           for (int r = g / CPR; r < kPairs; r += RPP) {
@@ -379,16 +375,16 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
 }
 
 int ret_fwd_pairs_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
-                     const int32_t* pairs, const int32_t* bsel, void* o_part, float* l_part, int* status, cudaStream_t st) {
-  const dim3 grid(d.Ck, rf::kSplit, d.B * d.Hq);
+                     const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st) {
+  const dim3 grid(d.k2 > 0 ? d.Ck * d.SB : d.Ck, rf::kSplit, d.B * d.Hq);     // one CTA (or a few) per key cluster, or per bucket
   prof_mark("k_ret_fwd_pairs_tc", st);
   if (d.D == 128) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_pairs_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, rf::Smem<128>::total));
-    k_ret_fwd_pairs_tc<128><<<grid, rf::kThreads, rf::Smem<128>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs, bsel,
+    k_ret_fwd_pairs_tc<128><<<grid, rf::kThreads, rf::Smem<128>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs,
                                                                           (bf16*)o_part, l_part, status);
   } else {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_fwd_pairs_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, rf::Smem<64>::total));
-    k_ret_fwd_pairs_tc<64><<<grid, rf::kThreads, rf::Smem<64>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs, bsel,
+    k_ret_fwd_pairs_tc<64><<<grid, rf::kThreads, rf::Smem<64>::total, st>>>(d, (const bf16*)Q, (const bf16*)Kp, (const bf16*)Vp, off_k, goff, pairs,
                                                                         (bf16*)o_part, l_part, status);
   }
   MUSE_LAUNCH_OK();
