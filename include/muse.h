@@ -248,6 +248,17 @@ MUSE_API long muse_profile_report(char* buf, size_t cap);
 MUSE_API int muse_test_force_paths(unsigned mask);
 MUSE_API int muse_test_wait_timeout(void* ws, unsigned limit_clocks, cudaStream_t stream);
 
+/* Bounds-checked build (no counterpart in the paper).  The same sources compiled with
+ * -DMUSE_DEBUG (python -m paper_2509_10406_b200.build --debug -> libmuse_debug.so) check every
+ * index that a kernel derives from data (assignments, selections, pair ids, bucket offsets,
+ * permutations) and the computed shared-memory offsets of its gathers against their bounds; an
+ * index out of range is recorded and the access skipped, nothing traps.  muse_debug_report waits
+ * for the device, writes one "file:line value v outside [0, n), c violation(s); " entry per source
+ * file that recorded one into text (HOST, text_bytes; may be NULL) and returns the number of such
+ * files, 0 when every check held; reset != 0 clears the records.  In the product build it
+ * returns MUSE_ERR_UNSUPPORTED.  Not thread-safe with respect to concurrent library calls. */
+MUSE_API int muse_debug_report(char* text, size_t text_bytes, int reset);
+
 /* Human-readable text for a return code (static storage). */
 MUSE_API const char* muse_strerror(int code);
 

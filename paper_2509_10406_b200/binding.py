@@ -14,7 +14,8 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libmuse.so")
+# MUSE_LIBRARY names another build of the same sources beside this file (the bounds-checked libmuse_debug.so)
+LIB_PATH = os.path.join(_HERE, os.path.basename(os.environ.get("MUSE_LIBRARY", "libmuse.so")))
 
 MUSE_BF16, MUSE_F32 = 0, 1
 MUSE_SEL_PER_QUERY, MUSE_SEL_PER_QCLUSTER = 0, 1
@@ -23,7 +24,7 @@ MUSE_INIT_INDICES, MUSE_INIT_STRIDED, MUSE_INIT_CENTRES = 0, 1, 2
 EXPORTS = ("muse_workspace_bytes", "muse_summaries_layout", "muse_cluster", "muse_summarize",
            "muse_attn_fwd", "muse_attn_bwd", "muse_cluster_noalloc", "muse_cluster_noalloc_max_bytes",
            "muse_cluster_noalloc_status_copy", "muse_status_copy", "muse_test_force_paths",
-           "muse_test_wait_timeout", "muse_profile", "muse_profile_report", "muse_strerror")
+           "muse_test_wait_timeout", "muse_debug_report", "muse_profile", "muse_profile_report", "muse_strerror")
 
 # bits of muse_test_force_paths
 FORCE_SUMM_FWD_SIMT, FORCE_FAR_SIMT, FORCE_SUMM_BWD_SIMT, FORCE_RET_FWD_STREAM = 1, 2, 4, 8
@@ -95,6 +96,7 @@ def lib() -> ctypes.CDLL:
         L.muse_status_copy.argtypes = [vp, vp, vp]
         L.muse_test_force_paths.argtypes = [ctypes.c_uint]
         L.muse_test_wait_timeout.argtypes = [vp, ctypes.c_uint, vp]
+        L.muse_debug_report.argtypes = [ctypes.c_char_p, sz, ctypes.c_int]
         L.muse_profile.argtypes = [ctypes.c_int]
         L.muse_profile_report.argtypes = [ctypes.c_char_p, sz]
         for name in EXPORTS[:-1]:
@@ -193,6 +195,13 @@ def muse_cluster_noalloc_status() -> int:
     out = torch.zeros(1, dtype=torch.int32, device="cuda")
     _check(lib().muse_cluster_noalloc_status_copy(_ptr(out), _stream()), "muse_cluster_noalloc_status_copy")
     return int(out.item())
+
+
+def muse_debug_report(reset: bool = True):
+    """(files with an out-of-range index, text) of a bounds-checked build; (MUSE_ERR_UNSUPPORTED, "") for the product build."""
+    buf = ctypes.create_string_buffer(4096)
+    n = lib().muse_debug_report(buf, 4096, int(reset))
+    return n, buf.value.decode()
 
 
 def muse_test_force_paths(mask: int) -> None:

@@ -1,6 +1,9 @@
 """Builds libmuse.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
 
-Usage: python -m paper_2509_10406_b200.build [--force] [--verbose]
+Usage: python -m paper_2509_10406_b200.build [--force] [--verbose] [--debug]
+
+--debug builds libmuse_debug.so instead: the same sources with -DMUSE_DEBUG (every data-derived index
+checked against its bound, violations recorded for muse_debug_report, nothing traps).
 """
 from __future__ import annotations
 
@@ -34,11 +37,14 @@ def _digest() -> str:
     return h.hexdigest()
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile every .cu under csrc/ and link libmuse.so; no-op when sources are unchanged."""
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Compile every .cu under csrc/ and link libmuse.so (libmuse_debug.so with debug); no-op when sources are unchanged."""
+    OBJ = os.path.join(CSRC, "build_debug" if debug else "build")
+    LIB = os.path.join(HERE, "libmuse_debug.so" if debug else "libmuse.so")
+    FLAGS = globals()["FLAGS"] + (["-DMUSE_DEBUG"] if debug else [])
     os.makedirs(OBJ, exist_ok=True)
     stamp = os.path.join(OBJ, "stamp")
-    dig = _digest()
+    dig = _digest() + ("-debug" if debug else "")
     if not force and os.path.exists(LIB) and os.path.exists(stamp) and open(stamp).read() == dig:
         return LIB
 
@@ -65,4 +71,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, debug="--debug" in sys.argv))

@@ -1,4 +1,5 @@
 // C-ABI entry points: argument validation on the host, then the stage launchers.
+#include <stdio.h>
 #include "common.cuh"
 #include "tc05.cuh"
 
@@ -68,7 +69,41 @@ int resolve(const muse_params_t* p, Dims* d) {
 
 namespace muse { bool path_forced(unsigned bit) { return (g_forced_paths & bit) != 0; } }
 
+#ifdef MUSE_DEBUG
+namespace muse {
+struct DbgEntry { const char* file; dbg_reader_t fn; };
+static DbgEntry g_dbg_tus[64];
+static int g_dbg_ntus = 0;
+void dbg_register(const char* file, dbg_reader_t fn) { if (g_dbg_ntus < 64) g_dbg_tus[g_dbg_ntus++] = DbgEntry{file, fn}; }
+}  // namespace muse
+#endif
+
 extern "C" {
+
+int muse_debug_report(char* text, size_t text_bytes, int reset) {
+  if (text != nullptr && text_bytes > 0) text[0] = 0;
+#ifdef MUSE_DEBUG
+  if (cudaDeviceSynchronize() != cudaSuccess) { cudaGetLastError(); return MUSE_ERR_CUDA; }
+  int bad = 0;
+  size_t used = 0;
+  for (int t = 0; t < muse::g_dbg_ntus; ++t) {
+    int rec[4];
+    muse::g_dbg_tus[t].fn(rec, reset);
+    if (rec[3] == 0) continue;
+    ++bad;
+    if (text != nullptr && used + 1 < text_bytes) {
+      const char* f = muse::g_dbg_tus[t].file;
+      for (const char* c = f; *c; ++c) if (*c == '/') f = c + 1;
+      const int w = snprintf(text + used, text_bytes - used, "%s:%d value %d outside [0, %d), %d violation(s); ", f, rec[0], rec[1], rec[2], rec[3]);
+      if (w > 0) used = used + (size_t)w < text_bytes ? used + (size_t)w : text_bytes - 1;
+    }
+  }
+  return bad;
+#else
+  (void)reset;
+  return MUSE_ERR_UNSUPPORTED;
+#endif
+}
 
 int muse_test_force_paths(unsigned mask) { g_forced_paths = mask; return MUSE_OK; }
 

@@ -616,6 +616,7 @@ __global__ void k_final_dkv(Dims dm, const int32_t* __restrict__ perm_k, const f
   if (e >= (long long)dm.N * (D / 4)) return;
   const int p = (int)(e / (D / 4)), q = (int)(e % (D / 4));
   const int u = perm_k[(size_t)pk * dm.N + p];
+  if (!MUSE_IN_RANGE(u, dm.N)) return;
   float4 ak = make_float4(0.f, 0.f, 0.f, 0.f), av = ak;
   for (int h = 0; h < dm.Hq; ++h) {
     if (dm.hm.g[h] != g) continue;

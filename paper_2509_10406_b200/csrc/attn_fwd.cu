@@ -74,7 +74,8 @@ __global__ void k_ret_fill(Dims d, const int32_t* __restrict__ sel, const int32_
     int base = 0;
     if (key >= 0 && lane == leader) base = atomicAdd(&cursor[(size_t)pq * d.SB * d.Ck + key], __popc(peers));
     base = __shfl_sync(0xffffffffu, base, leader);
-    if (key >= 0) pairs[(size_t)pq * npairs + base + __popc(peers & ((1u << lane) - 1u))] = pid;
+    if (key >= 0 && MUSE_IN_RANGE(base + __popc(peers & ((1u << lane) - 1u)), npairs))
+      pairs[(size_t)pq * npairs + base + __popc(peers & ((1u << lane) - 1u))] = pid;
   }
 }
 

@@ -25,6 +25,7 @@ k_block_select(Dims dm, const T* __restrict__ Q, const int32_t* __restrict__ ass
   const int pos = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (pos >= dm.N) return;
   const int t = perm_q[(size_t)pq * dm.N + pos];          // position in (block, query cluster) order -> query
+  if (!MUSE_IN_RANGE(t, dm.N)) return;
   const size_t row = (size_t)pq * dm.N + t;
   const int b = t / dm.Bs, m = dm.m, k2 = dm.k2;
   int32_t* bo = bsel_out + row * m * k2;
@@ -55,6 +56,7 @@ k_block_select(Dims dm, const T* __restrict__ Q, const int32_t* __restrict__ ass
     // block logits: lane b' ends up holding logit(b').  Lane b' fetches beta_b'; the rows are fetched four blocks at a
     // time so that their loads (and the four warp sums) are in flight together.
     const size_t e0 = ((size_t)pq * dm.SB * dm.Cq + i) * dm.Ck + j, estep = (size_t)dm.Cq * dm.Ck;   // entry of block 0, stride per block
+    if (!MUSE_IN_RANGE(e0 + (size_t)(b - 1) * estep, (size_t)gridDim.y * dm.SB * estep)) continue;
     const float be = lane < b ? sp.beta[e0 + lane * estep] : -INFINITY;
     const uint32_t live = __ballot_sync(0xffffffffu, be != -INFINITY);       // non-empty earlier blocks of the cluster
     float mine = -INFINITY;

@@ -145,7 +145,7 @@ k_sort_scatter(const int32_t* __restrict__ assign, int N, int C, int S, int Bs, 
         int rank = __popc(peers & ((1u << lane) - 1u));
         int start = live ? cur[key] : 0;
         __syncwarp();
-        if (live) {
+        if (live && MUSE_IN_RANGE(start + rank, N)) {
           pm[start + rank] = t;
           if (rank == __popc(peers) - 1) cur[key] = start + rank + 1;
         }
@@ -364,7 +364,10 @@ k_update(const T* __restrict__ X, int N, int C, int S, int kind, const int32_t* 
     for (int p = p0 + slot; p < p1; p += 4 * SLOTS) {
       int idx[4];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) idx[u] = p + u * SLOTS < p1 ? pm[p + u * SLOTS] : -1;
+      for (int u = 0; u < 4; ++u) {
+        idx[u] = p + u * SLOTS < p1 && MUSE_IN_RANGE(p + u * SLOTS, N) ? pm[p + u * SLOTS] : -1;
+        if (idx[u] >= 0 && !MUSE_IN_RANGE(idx[u], N)) idx[u] = -1;
+      }
       float v[4][VEC];
 #pragma unroll
       for (int u = 0; u < 4; ++u) {

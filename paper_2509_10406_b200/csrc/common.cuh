@@ -107,6 +107,31 @@ void prof_mark(const char* name, cudaStream_t st);
 constexpr int kStatusWords = 64;
 __device__ __forceinline__ void report_status(int* status, int code) { atomicCAS(status, 0, code); }
 
+// Bounds-checked build (compiled with -DMUSE_DEBUG into a second library): every index that a kernel derives from data
+// (assignments, selections, pair ids, bucket offsets, permutations) and the hand-computed shared-memory offsets of the
+// gathers pass through MUSE_IN_RANGE(index, bound).  A value outside [0, bound) is recorded (source line, value, bound,
+// count) in a per-source-file device record that muse_debug_report reads, and the caller skips the access: nothing
+// traps, the kernel runs to its end.  In the product build the macro is the constant `true` and the checks vanish.
+#ifdef MUSE_DEBUG
+static __device__ int g_dbg_rec[4];                      // {line, value, bound, violations} of this source file
+typedef void (*dbg_reader_t)(int out[4], int reset);
+void dbg_register(const char* file, dbg_reader_t fn);    // api.cu
+static void dbg_read_tu(int out[4], int reset) {
+  if (cudaMemcpyFromSymbol(out, g_dbg_rec, 16) != cudaSuccess) { out[0] = out[1] = out[2] = 0; out[3] = -1; cudaGetLastError(); }
+  if (reset) { const int z[4] = {0, 0, 0, 0}; if (cudaMemcpyToSymbol(g_dbg_rec, z, 16) != cudaSuccess) cudaGetLastError(); }
+}
+struct DbgReg { DbgReg() { dbg_register(__BASE_FILE__, &dbg_read_tu); } };
+static const DbgReg g_dbg_reg;
+__device__ __forceinline__ bool dbg_in_range(long long v, long long n, int line) {
+  if (v >= 0 && v < n) return true;
+  if (atomicAdd(&g_dbg_rec[3], 1) == 0) { g_dbg_rec[0] = line; g_dbg_rec[1] = (int)v; g_dbg_rec[2] = (int)n; }
+  return false;
+}
+#define MUSE_IN_RANGE(v, n) muse::dbg_in_range((long long)(v), (long long)(n), __LINE__)
+#else
+#define MUSE_IN_RANGE(v, n) true
+#endif
+
 // Test hook: bit set = take the library's other kernel for that step at shapes where the default is
 // the tensor-core kernel (muse_test_force_paths; never set in production).
 enum ForcePath : unsigned {

@@ -128,7 +128,8 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     // tile travels while the rows are gathered
     if (tid == ISSUER) { issue_kappa(0); issue_nu(0); }
     if (tid < NP * NR) {
-      const int t = tid < ns ? pm[s0 + tid] : -1;
+      int t = tid < ns && MUSE_IN_RANGE(s0 + tid, dm.N) ? pm[s0 + tid] : -1;
+      if (t >= 0 && !MUSE_IN_RANGE(t, dm.N)) t = -1;
       rows[tid] = t;
       Ls[tid] = t >= 0 ? LSE[(size_t)pq * dm.N + t] * kLog2e : 0.f;
       ds[tid] = t >= 0 ? delta[(size_t)pq * dm.N + t] : 0.f;
@@ -138,7 +139,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     for (int e = tid; e < NP * NR * CPR; e += THREADS) {
       const int r = e / CPR, ck = e % CPR, kb = ck >> 3, c = ck & 7, p = r / NR, rr = r % NR;
       uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
-      if (r < ns) {
+      if (r < ns && rows[r] >= 0) {
         a = reinterpret_cast<const uint4*>(Qp + (size_t)rows[r] * D)[ck];
         b = reinterpret_cast<const uint4*>(dOp + (size_t)rows[r] * D)[ck];
       }
@@ -147,7 +148,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     }
     for (int e = tid; e < ns * m; e += THREADS) {
       const int r = e / m, k = e % m;
-      const int c = sel[((size_t)pq * dm.N + rows[r]) * m + k];
+      const int c = rows[r] >= 0 ? sel[((size_t)pq * dm.N + rows[r]) * m + k] : -1;
       if (c >= 0 && c < Ck) atomicOr(&smask[2 * c + (r >> 5)], 1u << (r & 31));     // [cluster][row bits]
     }
     tc::fence_async_smem();
@@ -406,7 +407,7 @@ k_far_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
 #pragma unroll
           for (int r = 0; r < 32; ++r) {
             const int rr = p * NR + c0 + r;
-            if (rr < ns) atomicAdd(dQacc + ((size_t)pq * dm.N + rows[rr]) * D + L, v[r]);   // (result unused: no round trip)
+            if (rr < ns && rows[rr] >= 0) atomicAdd(dQacc + ((size_t)pq * dm.N + rows[rr]) * D + L, v[r]);   // (result unused: no round trip)
           }
         }
       }

@@ -329,7 +329,7 @@ k_far_fwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_khi, const __grid_c
     for (int e = tid; e < FR * (D / 8); e += NT) {
       const int r = e / (D / 8), ck = e % (D / 8), kb = ck >> 3, c = ck & 7;
       uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (r < n) v = reinterpret_cast<const uint4*>(Qp + (size_t)pm[r0 + r] * D)[ck];
+      if (r < n && MUSE_IN_RANGE(r0 + r, dm.N) && MUSE_IN_RANGE(pm[r0 + r], dm.N)) v = reinterpret_cast<const uint4*>(Qp + (size_t)pm[r0 + r] * D)[ck];
       *reinterpret_cast<uint4*>(Qs + kb * FR * 128 + tc::sw128_off(r, c)) = v;
     }
     tc::fence_async_smem();

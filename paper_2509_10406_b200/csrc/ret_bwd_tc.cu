@@ -143,11 +143,12 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
     for (int e = tid; e < kKeys * (D / 8); e += kThreads) {
       const int r = e / (D / 8), ck = e % (D / 8);
       uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
-      if (r < nkc) {
+      if (r < nkc && MUSE_IN_RANGE(k0 + kc + r, dm.N)) {
         a = reinterpret_cast<const uint4*>(Kb + (size_t)(kc + r) * D)[ck];
         b = reinterpret_cast<const uint4*>(Vb + (size_t)(kc + r) * D)[ck];
       }
       const uint32_t off = (ck >> 3) * kKeys * 128 + tc::sw128_off(r, ck & 7);
+      if (!MUSE_IN_RANGE(off, kKeys * D * 2 - 15)) continue;
       *reinterpret_cast<uint4*>(sm + oK + off) = a;
       *reinterpret_cast<uint4*>(sm + oV + off) = b;
     }
@@ -162,7 +163,8 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       // pair ids two tiles ahead and the rows' L, delta one tile ahead: no dependent global load at the top of a tile
       auto ld_pid = [&](int t) {
         const int t0 = g0 + t * kPairs;
-        return (t < ntiles && t0 + row < g1) ? __ldg(pr + t0 + row) : -1;
+        const int id = (t < ntiles && t0 + row < g1) ? __ldg(pr + t0 + row) : -1;
+        return id >= 0 && !MUSE_IN_RANGE(id, (long long)dm.N * dm.m) ? -1 : id;
       };
       int pid = ld_pid(tile0), pid_n = ld_pid(tile0 + tstep);
       float L2 = 0.f, dl = 0.f, L2_n = 0.f, dl_n = 0.f;
@@ -265,7 +267,7 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
             if (ok_) {
 #pragma unroll
               for (int u = 0; u < 32; ++u)
-                if (u0 + u < nkc) atomicAdd(dst + (size_t)(u0 + u) * D, x[u]);      // (result unused: no round trip)
+                if (u0 + u < nkc && MUSE_IN_RANGE(k0 + kc + u0 + u, dm.N)) atomicAdd(dst + (size_t)(u0 + u) * D, x[u]);      // (result unused: no round trip)
             }
           }
         }
@@ -344,6 +346,7 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
         for (int r = g / (D / 8); r < kPairs; r += RPP) {
           const int tok = tok_s[v][r];
           const size_t at = (size_t)max(tok, 0) * D + ck * 8;
+          if (!MUSE_IN_RANGE(tok + 1, dm.N + 1) || !MUSE_IN_RANGE((ck >> 3) * kPairs * 128 + tc::sw128_off(r, ck & 7), kPairs * D * 2 - 15)) continue;
           cp_async16(qd + tc::sw128_off(r, ck & 7), Qb + at, tok >= 0);
           cp_async16(od + tc::sw128_off(r, ck & 7), dOb + at, tok >= 0);
         }

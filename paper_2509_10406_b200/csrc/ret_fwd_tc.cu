@@ -143,11 +143,12 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
     for (int e = tid; e < kKeys * CPR; e += kThreads) {
       const int r = e / CPR, ck = e % CPR;
       uint4 a = make_uint4(0u, 0u, 0u, 0u), b = a;
-      if (kc + r < kall) {
+      if (kc + r < kall && MUSE_IN_RANGE(k0 + kc + r, dm.N)) {
         a = reinterpret_cast<const uint4*>(Kb + (size_t)(kc + r) * D)[ck];
         b = reinterpret_cast<const uint4*>(Vb + (size_t)(kc + r) * D)[ck];
       }
       const uint32_t off = (ck >> 3) * kKeys * 128 + tc::sw128_off(r, ck & 7);
+      if (!MUSE_IN_RANGE(off, kKeys * D * 2 - 15)) continue;
       *reinterpret_cast<uint4*>(sm + SM::k + off) = a;
       *reinterpret_cast<uint4*>(sm + SM::v + off) = b;
     }
@@ -164,6 +165,7 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       auto tile_ids = [&](int t, int& pid, int& last) {
         const int t0 = g0 + t * kPairs, nq = min(kPairs, g1 - t0);
         pid = (t < ntiles && row < nq) ? __ldg(pr + t0 + row) : -1;
+        if (pid >= 0 && !MUSE_IN_RANGE(pid, (long long)dm.N * mk)) pid = -1;
         last = t < ntiles ? __ldg(pr + t0 + nq - 1) : 0;
       };
       int pid, last;
@@ -347,6 +349,7 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
 #pragma unroll 4
           for (int r = g / CPR; r < kPairs; r += RPP) {
             const int tok = tok_s[r];
+            if (!MUSE_IN_RANGE(tok + 1, dm.N + 1) || !MUSE_IN_RANGE((ck >> 3) * kPairs * 128 + tc::sw128_off(r, ck & 7), kPairs * D * 2 - 15)) continue;
             cp_async16(qd + tc::sw128_off(r, ck & 7), Qb + (size_t)max(tok, 0) * D + ck * 8, tok >= 0);
           }
           asm volatile("cp.async.commit_group;" ::: "memory");

@@ -59,6 +59,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
   const int32_t* ok_ = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const int32_t* oq = off_q + (size_t)pq * (dm.S * dm.Cq + 1);
   const int kbeg = ok_[0];
+  (void)MUSE_IN_RANGE(ok_[dm.SB], dm.N + 1); (void)MUSE_IN_RANGE(kbeg, ok_[dm.SB] + 1);   // (the tiles come through tensor maps, which clip)
   if (kbeg >= ok_[dm.SB]) return;                       // no key of this cluster is ever summarised
   unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
   if (warp == 0) tc::tmem_alloc(&tbase_s, 512);

@@ -45,7 +45,9 @@ __global__ void k_gather_rows(const T* __restrict__ in, const int32_t* __restric
   const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= (long long)N * vpr) return;
   const int p = (int)(e / vpr), v = (int)(e % vpr);
-  const uint4* src = reinterpret_cast<const uint4*>(in + ((size_t)prob * N + perm[(size_t)prob * N + p]) * D);
+  const int t = perm[(size_t)prob * N + p];
+  if (!MUSE_IN_RANGE(t, N)) return;
+  const uint4* src = reinterpret_cast<const uint4*>(in + ((size_t)prob * N + t) * D);
   uint4* dst = reinterpret_cast<uint4*>(out + ((size_t)prob * N + p) * D);
   dst[v] = src[v];
 }
@@ -60,7 +62,7 @@ __global__ void k_bucket_sums(const T* __restrict__ Kp, const T* __restrict__ Vp
   const int bk = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (bk >= nbuckets) return;
   const int32_t* o = off_k + (size_t)prob * (nbuckets + 1) + bk;
-  const int p0 = o[0], p1 = o[1];
+  const int p0 = o[0], p1 = MUSE_IN_RANGE(o[1], N + 1) && MUSE_IN_RANGE(o[0], o[1] + 1) ? o[1] : o[0];
   constexpr int EPL = D / 32;
   float ak[EPL], av[EPL];
 #pragma unroll

@@ -123,6 +123,7 @@ k_summarize_tc(Dims dm, const __grid_constant__ CUtensorMap tm_K, const __grid_c
   if (tid == 32) issue_after(off[0]);
   for (int pl = 0; pl < dm.SB && ok; ++pl) {
     const int p0 = off[pl], p1 = off[pl + 1];
+    (void)MUSE_IN_RANGE(p1, dm.N + 1); (void)MUSE_IN_RANGE(p0, p1 + 1);     // (the tiles come through tensor maps, which clip)
     if (per_block) {                                     // the summary of block pl alone: the running state starts afresh
       M = -INFINITY; s = 0.f; T = 0.f;
 #pragma unroll

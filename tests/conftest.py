@@ -24,3 +24,15 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _bounds_checked_build_is_clean(request):
+    """When the suite runs against the bounds-checked build (MUSE_LIBRARY=libmuse_debug.so), no GPU test
+    may leave an out-of-range index on record."""
+    yield
+    if "gpu" not in request.keywords or "debug" not in os.environ.get("MUSE_LIBRARY", ""):
+        return
+    from paper_2509_10406_b200 import binding as mb
+    n, text = mb.muse_debug_report(reset=True)
+    assert n == 0, text
