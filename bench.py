@@ -274,9 +274,10 @@ def workload_config(w, gain):
 # DRAM bytes per (batch, head) problem from an ncu capture (--set full) of the headline workload cut
 # to one head: dram__bytes_read.sum + dram__bytes_write.sum per launch.  Traffic grows in proportion
 # to the problem count.
-NCU_TRAFFIC_PER_HEAD = {"k_summarize_tc": 1.430e9, "k_local_fwd_tc": 0.056e9, "k_far_fwd_tc": 1.634e9,
-                        "k_ret_bwd_fused_tc": 0.608e9, "k_ret_fwd_cluster_tc": 0.529e9, "k_far_bwd_tc": 2.411e9,
-                        "k_summ_bwd_tc": 1.102e9, "k_local_bwd_dkdv_tc": 0.088e9, "k_local_bwd_dq_tc": 0.073e9}
+NCU_TRAFFIC_PER_HEAD = {"k_summarize_tc": 1.430e9, "k_local_fwd_tc": 0.055e9, "k_far_fwd_tc": 1.630e9,
+                        "k_ret_bwd_pairs_tc": 1.235e9, "k_ret_fwd_pairs_tc": 0.498e9, "k_far_bwd_tc": 2.415e9,
+                        "k_summ_bwd_tc": 1.100e9, "k_local_bwd_dkdv_tc": 0.087e9, "k_local_bwd_dq_tc": 0.074e9,
+                        "k_merge": 0.566e9, "k_final_dq": 0.528e9}
 
 
 def main():
