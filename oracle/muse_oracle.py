@@ -37,7 +37,10 @@ reproduces k2 = all; a separately written single softmax over exact and stand-in
 inputs; singleton key or query clusters stay exact for every k2; weights causal, sum to one.  Dipole: the Jacobian
 of the far field at zero residual equals the dense-attention Jacobian (a
 cross-covariance written separately in the test), the error falls from first
-to second order in the residual, causality and key-translation invariance.
+to second order in the residual, causality and key-translation invariance.  Streaming k-means: closed-form
+exponentially weighted means for one cluster and for separated blobs, a hand-computed case that tells
+minibatch assignment from immediate updates, continuation from a saved state; balanced assignment: equals
+the nearest centroid when the cap does not bind, hand-computed overflow cases, size and placement invariants.
 """
 from __future__ import annotations
 
@@ -48,6 +51,7 @@ __all__ = [
     "block_summaries", "accumulate", "accumulated_summaries",
     "select_clusters", "forward", "backward", "layer_forward", "layer_backward",
     "untilted_covariances", "merged_dipole",
+    "stream_order", "streaming_kmeans", "balanced_cap", "balanced_assign",
 ]
 
 _M64 = (1 << 64) - 1
@@ -133,6 +137,87 @@ def strided_init(N: int, C: int, seed: int, stream: int) -> np.ndarray:
     bijection above: index r -> position pi(r * floor(N/C))."""
     stride = N // C
     return np.array([feistel_permute(r * stride, N, seed, stream) for r in range(C)], np.int32)
+
+
+# --------------------------------------------------------------------------------------------
+# The paper's own clustering (Appendix "Clustering Details": "Centroid Computation",
+# "Balanced Assignment"): one pass of streaming mini-batch k-means, then a per-block assignment
+# under a size cap.  Readings where the appendix is silent: the stream visits the vectors in the
+# order of the seeded shuffle (position s of the stream is vector pi(s)); centroid r starts as
+# the r-th strided sample with total t = x and count c = 1; a minibatch is assigned against the
+# centroids as they stand when it starts, then its updates are applied one vector after the
+# other; the cap is ceil(factor * B / K) per (block, cluster); a vector that loses its nearest
+# centroid to the cap is placed by the two-step rule stated at balanced_assign.  Arithmetic in
+# fp64 here (the paper runs it in half precision for speed; nothing in the method depends on that).
+# --------------------------------------------------------------------------------------------
+
+def stream_order(N: int, seed: int, stream: int) -> np.ndarray:
+    """The shuffled visiting order of the single pass: position s -> vector pi(s)."""
+    return np.array([feistel_permute(s, N, seed, stream) for s in range(N)], np.int64)
+
+
+def streaming_kmeans(X, C, order, init_idx, batch=64, beta=0.9, first_batch=0, n_batches=None,
+                     totals=None, counts=None):
+    """Appendix "Centroid Computation", step 2.  For each minibatch of `batch` vectors of the
+    stream: assign every vector to its nearest current centroid t_j / c_j, then for each vector x
+    in stream order t_j <- beta t_j + x, c_j <- beta c_j + 1 for its centroid j.  Runs minibatches
+    [first_batch, first_batch + n_batches) from the given state (first_batch = 0: the start state
+    t = X[init_idx], c = 1).  Returns (centres, totals, counts, assignments of the streamed vectors)."""
+    X = np.asarray(X, np.float64)
+    N = X.shape[0]
+    nb_all = (N + batch - 1) // batch
+    if n_batches is None:
+        n_batches = nb_all - first_batch
+    if totals is None:
+        totals = X[np.asarray(init_idx, np.int64)].copy()
+        counts = np.ones(C)
+    else:
+        totals, counts = np.array(totals, np.float64, copy=True), np.array(counts, np.float64, copy=True)
+    seen = []
+    for s in range(first_batch, first_batch + n_batches):
+        idx = np.asarray(order[s * batch:min(N, (s + 1) * batch)], np.int64)
+        a = assign_nearest(X[idx], totals / counts[:, None])
+        for u, j in zip(idx, a):
+            totals[j] = beta * totals[j] + X[u]
+            counts[j] = beta * counts[j] + 1.0
+        seen.append(a)
+    return totals / counts[:, None], totals, counts, (np.concatenate(seen) if seen else np.zeros(0, np.int32))
+
+
+def balanced_cap(Bs: int, C: int, factor: float) -> int:
+    """Largest allowed size of a (block, cluster) bucket: factor x the average B / K, rounded up."""
+    return int(np.ceil(factor * Bs / C))
+
+
+def balanced_assign(X, centres, S, factor=4.0):
+    """Appendix "Balanced Assignment": independently in each spatial block, every vector goes to its
+    nearest centroid subject to a maximum bucket size.  Step 1: every vector names its nearest
+    centroid; of the vectors of a block that name centroid j, the first cap in position order keep it.
+    Step 2: the others, in position order, take the nearest centroid whose bucket still has room
+    (counting the step-1 members and the step-2 vectors placed before).  Ties -> lowest centroid."""
+    X = np.asarray(X, np.float64)
+    centres = np.asarray(centres, np.float64)
+    N, C = X.shape[0], centres.shape[0]
+    Bs = N // S
+    cap = balanced_cap(Bs, C, factor)
+    d = (centres * centres).sum(1)[None, :] - 2.0 * (X @ centres.T)
+    out = np.full(N, -1, np.int32)
+    for b in range(S):
+        size = np.zeros(C, np.int64)
+        late = []
+        for t in range(b * Bs, (b + 1) * Bs):
+            j = int(np.argmin(d[t]))
+            if size[j] < cap:
+                out[t] = j
+                size[j] += 1
+            else:
+                late.append(t)
+        for t in late:
+            dd = np.where(size < cap, d[t], np.inf)
+            j = int(np.argmin(dd))
+            out[t] = j
+            size[j] += 1
+    return out
 
 
 # --------------------------------------------------------------------------------------------

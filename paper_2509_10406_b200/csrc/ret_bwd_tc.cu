@@ -178,6 +178,11 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       for (int tile = tile0; tile < ntiles; tile += tstep, ++np) {
         const int pid_nn = ld_pid(tile + 2 * tstep);
         ld_scalars(pid_n, L2_n, dl_n);
+        if (!first && pid_n >= 0) {                         // a later sweep adds to the stored dQ row: have the next tile's row on its way
+          const char* pf = reinterpret_cast<const char*>(dq_part + (pbase + pid_n) * D);
+#pragma unroll
+          for (int o = 0; o < D * 2; o += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(pf + o));
+        }
         const int vis = pid >= 0 ? visible(pid, kc) : 0;
         const uint32_t ph = np & 1;
         RBCLK(0)

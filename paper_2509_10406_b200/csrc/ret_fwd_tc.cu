@@ -173,6 +173,12 @@ k_ret_fwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       for (; tile < ntiles; tile += nsub) {
         int pid_n, last_n;
         tile_ids(tile + nsub, pid_n, last_n);
+        if (!first && pid_n >= 0) {                         // a later sweep merges into the stored row: have the next tile's row on its way
+          const char* pf = reinterpret_cast<const char*>(o_part + (pbase + pid_n) * D);
+#pragma unroll
+          for (int o = 0; o < D * 2; o += 128) asm volatile("prefetch.global.L2 [%0];" ::"l"(pf + o));
+          asm volatile("prefetch.global.L2 [%0];" ::"l"(l_part + pbase + pid_n));
+        }
         const int nk = visible(last, kc), nk16 = (nk + 15) & ~15;      // the tile's last pair has the latest plane: it sees the most keys
         // which of the sweep's 128 key columns this row sees (a prefix: the cluster's keys of the earlier blocks, or the bucket)
         uint32_t vm[4] = {0u, 0u, 0u, 0u};
