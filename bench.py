@@ -297,6 +297,9 @@ def main():
     ap.add_argument("--forward-only", action="store_true", help="time cluster + summarize + forward only")
     ap.add_argument("--k2", type=int, default=0,
                     help="spatial blocks retrieved inside each selected cluster (0 = all; > 0 is forward only)")
+    ap.add_argument("--clustering", default="lloyd", choices=["lloyd", "streaming"],
+                    help="lloyd = muse_cluster (the measured path); streaming = the paper's one-pass mini-batch k-means "
+                         "with the balanced per-block assignment (muse_cluster_streaming; device-timed line only)")
     ap.add_argument("--dipole", action="store_true",
                     help="far field with the dipole correction instead of retrieval (sets m = 0, forward only)")
     ap.add_argument("--ref-rows", type=int, default=128, help="sampled queries for the oracle timing")
@@ -315,6 +318,9 @@ def main():
         args.forward_only = True
     if args.k2 > 0:
         args.forward_only = True
+    if args.clustering == "streaming":                    # a device-timed comparison line: no staged run, no oracle sample
+        args.no_e2e = True
+        args.no_cpu_baseline = True
     if args.kmeans_iters is not None:
         w = w.with_(T=args.kmeans_iters)
     if args.heads is not None:
@@ -358,6 +364,8 @@ def main():
     p = mb.make_params(B=w.B, Hq=hq, Hkv=hkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=w.m, n_blocks=w.S,
                        dtype=w.dtype, kmeans_iters=w.T, dipole=int(args.dipole), k2=args.k2)
     buf = mb.MuseBuffers(p, backward=not args.forward_only)
+    stream_ws = (torch.zeros(mb.muse_stream_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+                 if args.clustering == "streaming" else None)
     O_all = torch.empty_like(Q)
     dQ_all, dK_all, dV_all = (None, None, None) if args.forward_only else (torch.empty_like(Q), torch.empty_like(K), torch.empty_like(V))
 
@@ -371,7 +379,10 @@ def main():
         for g in range(groups):
             qs, ks = slice(g * hq, (g + 1) * hq), slice(g * hkv, (g + 1) * hkv)
             Qg, Kg, Vg = Q[:, qs], K[:, ks], V[:, ks]
-            mb.muse_cluster(p, Qg, Kg, init_q[:, qs], init_k[:, ks], buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, buf.ws)
+            if args.clustering == "streaming":
+                mb.muse_cluster_streaming(p, Qg, Kg, buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, stream_ws, beta=0.9, cap_factor=4.0)
+            else:
+                mb.muse_cluster(p, Qg, Kg, init_q[:, qs], init_k[:, ks], buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, buf.ws)
             m_("cluster")
             mb.muse_summarize(p, Kg, Vg, buf.assign_k, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
             m_("summarize")
@@ -617,6 +628,27 @@ def main():
             del bd
         except Exception as ex:
             context["dense_own_kernels_error"] = repr(ex)[:200]
+    if args.clustering == "streaming":
+        # quality beside the time: the k-means objective (mean squared distance to the assigned centroid, head 0 of the
+        # last head group) under the streaming pass + balanced assignment and under Lloyd, and how many vectors the cap
+        # moved away from their nearest centroid.  Bench-only arithmetic (torch), outside every timed region.
+        def objective(X, a, c):
+            return float(((X.float() - c[a.long()]) ** 2).sum(-1).mean().item())
+        g0 = groups - 1
+        Qg, Kg = Q[:, g0 * hq:(g0 + 1) * hq], K[:, g0 * hkv:(g0 + 1) * hkv]
+        qual = {"streaming_objective_q": objective(Qg[0, 0], buf.assign_q[0, 0], buf.qbar[0, 0]),
+                "streaming_objective_k": objective(Kg[0, 0], buf.assign_k[0, 0], buf.kcent[0, 0])}
+        near = torch.empty_like(buf.assign_k)
+        mb.muse_balanced_assign(p, Kg, 1, buf.kcent, near, stream_ws, cap_factor=0.0)
+        qual["keys_moved_by_the_cap_fraction"] = float((near != buf.assign_k).float().mean().item())
+        nearq = torch.empty_like(buf.assign_q)
+        mb.muse_balanced_assign(p, Qg, 0, buf.qbar, nearq, stream_ws, cap_factor=0.0)
+        qual["queries_moved_by_the_cap_fraction"] = float((nearq != buf.assign_q).float().mean().item())
+        mb.muse_cluster(p, Qg, Kg, init_q[:, g0 * hq:(g0 + 1) * hq], init_k[:, g0 * hkv:(g0 + 1) * hkv], buf.assign_q, buf.assign_k,
+                        buf.qbar, buf.kcent, buf.ws)
+        qual["lloyd_objective_q"] = objective(Qg[0, 0], buf.assign_q[0, 0], buf.qbar[0, 0])
+        qual["lloyd_objective_k"] = objective(Kg[0, 0], buf.assign_k[0, 0], buf.kcent[0, 0])
+        context["clustering_quality_head0"] = qual
     if not args.no_sharp and args.gain == 1.0:
         # the same step on the sharp variant of the inputs (Q x 128, exact in bf16): attention is then peaked,
         # so selection and retrieval matter; k-means and the tile schedule are scale-free
@@ -645,7 +677,9 @@ def main():
             "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": w.dtype,
             "data": "synthetic",
             "config": dict(workload_config(w, args.gain), head_stages=groups,
-                           dipole=int(args.dipole), k2=args.k2, passes="cluster+summarize+forward" if args.forward_only else "cluster+summarize+forward+backward"),
+                           dipole=int(args.dipole), k2=args.k2,
+                           clustering="lloyd" if args.clustering == "lloyd" else "streaming mini-batch k-means (batch 64, beta 0.9) + balanced assignment (cap 4 B/K)",
+                           passes="cluster+summarize+forward" if args.forward_only else "cluster+summarize+forward+backward"),
             "ms_per_step_median": statistics.median(per_step), "ms_per_step_best": min(per_step), "stages_ms": stages,
             "clocks": clocks, "e2e": e2e,
             "gpu_launches": launches, "roofline": roof, "cpu_baseline": cpu, "kernels": kernels, "context": context,

@@ -227,6 +227,46 @@ MUSE_API int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K,
                   const int32_t* sel, void* dQ, void* dK, void* dV,
                   void* ws, size_t ws_bytes, cudaStream_t stream);
 
+/* The paper's own clustering (Appendix "Clustering Details").  An alternative to muse_cluster with the
+ * same outputs; the rest of the path does not care which produced them.
+ *
+ * muse_stream_kmeans - "Centroid Computation": ONE pass of streaming mini-batch k-means over the vectors X
+ *   (DEVICE, [B,Hq,N,D] for side 0 = queries with C_q centroids, [B,Hkv,N,D] for side 1 = keys with C_k) of
+ *   every head.  The vectors are visited in the order of the seeded shuffle (p->seed; the same bijection as
+ *   MUSE_INIT_STRIDED, position s of the stream = vector pi(s)), MUSE_STREAM_BATCH = 64 per minibatch; a
+ *   minibatch is assigned to the nearest current centroids t_j / c_j (|c|^2 - 2 x.c, ties to the lower
+ *   index), then its vectors update their centroids one after the other in stream order:
+ *   t_j <- beta t_j + x, c_j <- beta c_j + 1 (the paper uses beta = 0.9).  Centroid r starts as the r-th
+ *   strided sample of the shuffled sequence with t = x, c = 1.  The call runs minibatches
+ *   [first_batch, first_batch + n_batches) (n_batches < 0: up to the last, which may be short):
+ *   first_batch = 0 starts from the start state, otherwise from the state in totals / counts.
+ *   totals [problems, C, D] fp32 and counts [problems, C] fp32 (DEVICE, in/out: the state t, c),
+ *   centres [problems, C, D] fp32 (DEVICE, out: t_j / c_j), assign_stream [problems, N] int32 (DEVICE, out,
+ *   may be NULL: the centroid each streamed vector was assigned to, by stream position; positions outside
+ *   the call's minibatches are not written).  fp32 arithmetic.  ws: >= 256 bytes (status words only).
+ * muse_balanced_assign - "Balanced Assignment": independently in each spatial block, every vector goes to
+ *   its nearest centroid subject to a bucket size of at most cap = ceil(cap_factor * B / K) (the paper uses
+ *   cap_factor = 4).  The paper gives no rule for a vector whose nearest centroid is full; the one taken:
+ *   (1) every vector names its nearest centroid, and of the vectors of a block that name centroid j the
+ *   first cap in position order keep it; (2) the others, in position order, take the nearest centroid
+ *   whose bucket still has room (counting step-1 members and earlier step-2 placements).  cap_factor <= 0:
+ *   no cap (plain nearest centroid).  centres [problems, C, D] fp32 (DEVICE, in), assign [problems, N]
+ *   int32 (DEVICE, out).  ws: muse_stream_workspace_bytes.
+ * muse_cluster_streaming - both steps for Q and/or K (either may be NULL with its outputs), with the
+ *   streaming state kept in ws; outputs as muse_cluster.  ws: muse_stream_workspace_bytes.
+ * Errors as for muse_cluster; beta outside (0, 1] is MUSE_ERR_INVALID_ARG. */
+#define MUSE_STREAM_BATCH 64
+MUSE_API int muse_stream_workspace_bytes(const muse_params_t* p, size_t* bytes);
+MUSE_API int muse_stream_kmeans(const muse_params_t* p, const void* X, int side, float beta, int first_batch,
+                                int n_batches, float* totals, float* counts, float* centres,
+                                int32_t* assign_stream, void* ws, size_t ws_bytes, cudaStream_t stream);
+MUSE_API int muse_balanced_assign(const muse_params_t* p, const void* X, int side, const float* centres,
+                                  float cap_factor, int32_t* assign, void* ws, size_t ws_bytes,
+                                  cudaStream_t stream);
+MUSE_API int muse_cluster_streaming(const muse_params_t* p, const void* Q, const void* K, float beta,
+                                    float cap_factor, int32_t* assign_q, int32_t* assign_k, float* qbar,
+                                    float* kcent, void* ws, size_t ws_bytes, cudaStream_t stream);
+
 /* Per-kernel timing for benchmarks (no counterpart in the paper).  muse_profile(1) clears the
  * record and makes every later library call record CUDA events on its stream around each
  * kernel launch (events are created on demand and reused); muse_profile(0) stops recording.

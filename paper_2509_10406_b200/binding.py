@@ -22,7 +22,8 @@ MUSE_SEL_PER_QUERY, MUSE_SEL_PER_QCLUSTER = 0, 1
 MUSE_INIT_INDICES, MUSE_INIT_STRIDED, MUSE_INIT_CENTRES = 0, 1, 2
 
 EXPORTS = ("muse_workspace_bytes", "muse_summaries_layout", "muse_cluster", "muse_summarize",
-           "muse_attn_fwd", "muse_attn_bwd", "muse_cluster_noalloc", "muse_cluster_noalloc_max_bytes",
+           "muse_attn_fwd", "muse_attn_bwd", "muse_stream_workspace_bytes", "muse_stream_kmeans", "muse_balanced_assign",
+           "muse_cluster_streaming", "muse_cluster_noalloc", "muse_cluster_noalloc_max_bytes",
            "muse_cluster_noalloc_status_copy", "muse_status_copy", "muse_test_force_paths",
            "muse_test_wait_timeout", "muse_debug_report", "muse_profile", "muse_profile_report", "muse_strerror")
 
@@ -90,6 +91,11 @@ def lib() -> ctypes.CDLL:
         L.muse_attn_fwd.argtypes = [pp, vp, vp, vp, i32p, f32p, i32p, i32p, vp, i32p, i32p, vp, f32p, i32p, i32p, vp, sz, vp]
         L.muse_attn_bwd.argtypes = [pp, vp, vp, vp, vp, f32p, vp, i32p, f32p, i32p, i32p, vp, i32p, vp, vp, vp,
                                     vp, sz, vp]
+        fl, ci = ctypes.c_float, ctypes.c_int
+        L.muse_stream_workspace_bytes.argtypes = [pp, ctypes.POINTER(sz)]
+        L.muse_stream_kmeans.argtypes = [pp, vp, ci, fl, ci, ci, f32p, f32p, f32p, i32p, vp, sz, vp]
+        L.muse_balanced_assign.argtypes = [pp, vp, ci, f32p, fl, i32p, vp, sz, vp]
+        L.muse_cluster_streaming.argtypes = [pp, vp, vp, fl, fl, i32p, i32p, f32p, f32p, vp, sz, vp]
         L.muse_cluster_noalloc.argtypes = [pp, vp, vp, i32p, i32p, i32p, i32p, f32p, f32p, vp]
         L.muse_cluster_noalloc_max_bytes.argtypes = []
         L.muse_cluster_noalloc_status_copy.argtypes = [vp, vp]
@@ -189,6 +195,29 @@ def muse_status(ws) -> int:
     out = torch.zeros(1, dtype=torch.int32, device=ws.device)
     _check(lib().muse_status_copy(_ptr(ws), _ptr(out), _stream()), "muse_status_copy")
     return int(out.item())
+
+
+def muse_stream_workspace_bytes(p) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().muse_stream_workspace_bytes(ctypes.byref(p), ctypes.byref(out)), "muse_stream_workspace_bytes")
+    return int(out.value)
+
+
+def muse_stream_kmeans(p, X, side, totals, counts, centres, ws, beta=0.9, first_batch=0, n_batches=-1, assign_stream=None):
+    _check(lib().muse_stream_kmeans(ctypes.byref(p), _ptr(X), int(side), float(beta), int(first_batch), int(n_batches),
+                                    _ptr(totals), _ptr(counts), _ptr(centres), _ptr(assign_stream), _ptr(ws),
+                                    ws.numel() * ws.element_size(), _stream()), "muse_stream_kmeans")
+
+
+def muse_balanced_assign(p, X, side, centres, assign, ws, cap_factor=4.0):
+    _check(lib().muse_balanced_assign(ctypes.byref(p), _ptr(X), int(side), _ptr(centres), float(cap_factor), _ptr(assign),
+                                      _ptr(ws), ws.numel() * ws.element_size(), _stream()), "muse_balanced_assign")
+
+
+def muse_cluster_streaming(p, Q, K, assign_q, assign_k, qbar, kcent, ws, beta=0.9, cap_factor=4.0):
+    _check(lib().muse_cluster_streaming(ctypes.byref(p), _ptr(Q), _ptr(K), float(beta), float(cap_factor), _ptr(assign_q),
+                                        _ptr(assign_k), _ptr(qbar), _ptr(kcent), _ptr(ws), ws.numel() * ws.element_size(),
+                                        _stream()), "muse_cluster_streaming")
 
 
 def muse_cluster_noalloc_status() -> int:

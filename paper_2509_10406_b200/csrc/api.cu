@@ -1,5 +1,6 @@
 // C-ABI entry points: argument validation on the host, then the stage launchers.
 #include <stdio.h>
+#include <algorithm>
 #include "common.cuh"
 #include "tc05.cuh"
 
@@ -181,6 +182,85 @@ int muse_cluster(const muse_params_t* p, const void* Q, const void* K, const int
     if (assign_k == nullptr || kcent == nullptr || !aligned16(K) || !aligned16(kcent)) return MUSE_ERR_INVALID_ARG;
     if (p->init_mode == MUSE_INIT_INDICES && init_k == nullptr) return MUSE_ERR_INVALID_ARG;
     rc = lloyd(d, p->dtype, K, d.B * d.Hkv, d.Ck, 1, init_k, p->init_mode, p->seed, p->kmeans_iters, assign_k, kcent, ws, stream);
+    if (rc != MUSE_OK) return rc;
+  }
+  prof_mark(nullptr, stream);
+  return MUSE_OK;
+}
+
+static size_t up256(size_t x) { return (x + 255) & ~size_t(255); }
+
+int muse_stream_workspace_bytes(const muse_params_t* p, size_t* bytes) {
+  Dims d;
+  int rc = resolve(p, &d);
+  if (rc != MUSE_OK) return rc;
+  if (bytes == nullptr) return MUSE_ERR_INVALID_ARG;
+  const size_t pq = (size_t)d.B * d.Hq, pk = (size_t)d.B * d.Hkv;
+  const size_t bal = std::max(balanced_ws_bytes(d, (int)pq, d.Cq), balanced_ws_bytes(d, (int)pk, d.Ck));
+  const size_t tot = std::max(pq * d.Cq, pk * d.Ck);
+  *bytes = up256(bal) + up256(tot * d.D * sizeof(float)) + up256(tot * sizeof(float));
+  return MUSE_OK;
+}
+
+int muse_stream_kmeans(const muse_params_t* p, const void* X, int side, float beta, int first_batch, int n_batches,
+                       float* totals, float* counts, float* centres, int32_t* assign_stream, void* ws, size_t ws_bytes,
+                       cudaStream_t stream) {
+  Dims d;
+  int rc = resolve(p, &d);
+  if (rc != MUSE_OK) return rc;
+  if (!X || !totals || !counts || !centres || !ws || (side != 0 && side != 1)) return MUSE_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(totals) || !aligned16(centres) || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;
+  if (!(beta > 0.f) || beta > 1.f) return MUSE_ERR_INVALID_ARG;
+  if (ws_bytes < 256) return MUSE_ERR_WORKSPACE;
+  if (clear_status(ws, stream) != MUSE_OK) return MUSE_ERR_CUDA;
+  rc = stream_kmeans(d, p->dtype, X, side == 0 ? d.B * d.Hq : d.B * d.Hkv, side == 0 ? d.Cq : d.Ck, side, p->seed, beta,
+                     first_batch, n_batches, totals, counts, centres, assign_stream, stream);
+  prof_mark(nullptr, stream);
+  return rc;
+}
+
+int muse_balanced_assign(const muse_params_t* p, const void* X, int side, const float* centres, float cap_factor,
+                         int32_t* assign, void* ws, size_t ws_bytes, cudaStream_t stream) {
+  Dims d;
+  int rc = resolve(p, &d);
+  if (rc != MUSE_OK) return rc;
+  if (!X || !centres || !assign || !ws || (side != 0 && side != 1)) return MUSE_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(centres) || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;
+  const int problems = side == 0 ? d.B * d.Hq : d.B * d.Hkv, C = side == 0 ? d.Cq : d.Ck;
+  if (ws_bytes < balanced_ws_bytes(d, problems, C)) return MUSE_ERR_WORKSPACE;
+  if (clear_status(ws, stream) != MUSE_OK) return MUSE_ERR_CUDA;
+  rc = balanced_assign(d, p->dtype, X, problems, C, side, centres, cap_factor, assign, ws, stream);
+  prof_mark(nullptr, stream);
+  return rc;
+}
+
+int muse_cluster_streaming(const muse_params_t* p, const void* Q, const void* K, float beta, float cap_factor,
+                           int32_t* assign_q, int32_t* assign_k, float* qbar, float* kcent, void* ws, size_t ws_bytes,
+                           cudaStream_t stream) {
+  Dims d;
+  int rc = resolve(p, &d);
+  if (rc != MUSE_OK) return rc;
+  if (ws == nullptr || !aligned16(ws) || (Q == nullptr && K == nullptr)) return MUSE_ERR_INVALID_ARG;
+  if (!(beta > 0.f) || beta > 1.f) return MUSE_ERR_INVALID_ARG;
+  size_t need = 0;
+  muse_stream_workspace_bytes(p, &need);
+  if (ws_bytes < need) return MUSE_ERR_WORKSPACE;
+  if (clear_status(ws, stream) != MUSE_OK) return MUSE_ERR_CUDA;
+  const size_t pq = (size_t)d.B * d.Hq, pk = (size_t)d.B * d.Hkv;
+  const size_t bal = up256(std::max(balanced_ws_bytes(d, (int)pq, d.Cq), balanced_ws_bytes(d, (int)pk, d.Ck)));
+  const size_t tot = std::max(pq * d.Cq, pk * d.Ck);
+  float* totals = reinterpret_cast<float*>((char*)ws + bal);
+  float* counts = reinterpret_cast<float*>((char*)ws + bal + up256(tot * d.D * sizeof(float)));
+  for (int side = 0; side < 2; ++side) {
+    const void* X = side == 0 ? Q : K;
+    if (X == nullptr) continue;
+    int32_t* assign = side == 0 ? assign_q : assign_k;
+    float* cen = side == 0 ? qbar : kcent;
+    if (assign == nullptr || cen == nullptr || !aligned16(X) || !aligned16(cen)) return MUSE_ERR_INVALID_ARG;
+    const int problems = side == 0 ? (int)pq : (int)pk, C = side == 0 ? d.Cq : d.Ck;
+    rc = stream_kmeans(d, p->dtype, X, problems, C, side, p->seed, beta, 0, -1, totals, counts, cen, nullptr, stream);
+    if (rc != MUSE_OK) return rc;
+    rc = balanced_assign(d, p->dtype, X, problems, C, side, cen, cap_factor, assign, ws, stream);
     if (rc != MUSE_OK) return rc;
   }
   prof_mark(nullptr, stream);

@@ -151,6 +151,15 @@ int lloyd(const Dims& d, int dtype, const void* X, int problems, int C, int kind
           int32_t* assign, float* centres, void* ws, cudaStream_t st);
 size_t lloyd_ws_bytes(const Dims& d, int problems, int C, int kind);
 
+// the paper's own clustering: one streaming pass (state = totals, counts; n_batches < 0: to the end) and the
+// per-block assignment under a bucket-size cap (factor <= 0: plain nearest centroid)
+int stream_kmeans(const Dims& d, int dtype, const void* X, int problems, int C, int kind, uint64_t seed, float beta,
+                  int first_batch, int n_batches, float* totals, float* counts, float* centres, int32_t* assign_stream,
+                  cudaStream_t st);
+int balanced_assign(const Dims& d, int dtype, const void* X, int problems, int C, int kind, const float* centres, float factor,
+                    int32_t* assign, void* ws, cudaStream_t st);
+size_t balanced_ws_bytes(const Dims& d, int problems, int C);
+
 // assign_k == nullptr: the keys are already bucketed (off_k, perm_k are inputs) and `status` names the
 // caller's status words; counts / ksum / vsum (untilted per-bucket statistics) may be nullptr
 int summarize(const Dims& d, int dtype, const void* K, const void* V, const int32_t* assign_k,
