@@ -214,7 +214,7 @@ int muse_stream_kmeans(const muse_params_t* p, const void* X, int side, float be
   if (ws_bytes < 256) return MUSE_ERR_WORKSPACE;
   if (clear_status(ws, stream) != MUSE_OK) return MUSE_ERR_CUDA;
   rc = stream_kmeans(d, p->dtype, X, side == 0 ? d.B * d.Hq : d.B * d.Hkv, side == 0 ? d.Cq : d.Ck, side, p->seed, beta,
-                     first_batch, n_batches, totals, counts, centres, assign_stream, stream);
+                     first_batch, n_batches, totals, counts, centres, assign_stream, (int32_t*)ws, stream);
   prof_mark(nullptr, stream);
   return rc;
 }
@@ -258,7 +258,7 @@ int muse_cluster_streaming(const muse_params_t* p, const void* Q, const void* K,
     float* cen = side == 0 ? qbar : kcent;
     if (assign == nullptr || cen == nullptr || !aligned16(X) || !aligned16(cen)) return MUSE_ERR_INVALID_ARG;
     const int problems = side == 0 ? (int)pq : (int)pk, C = side == 0 ? d.Cq : d.Ck;
-    rc = stream_kmeans(d, p->dtype, X, problems, C, side, p->seed, beta, 0, -1, totals, counts, cen, nullptr, stream);
+    rc = stream_kmeans(d, p->dtype, X, problems, C, side, p->seed, beta, 0, -1, totals, counts, cen, nullptr, (int32_t*)ws, stream);
     if (rc != MUSE_OK) return rc;
     rc = balanced_assign(d, p->dtype, X, problems, C, side, cen, cap_factor, assign, ws, stream);
     if (rc != MUSE_OK) return rc;

@@ -155,7 +155,7 @@ size_t lloyd_ws_bytes(const Dims& d, int problems, int C, int kind);
 // per-block assignment under a bucket-size cap (factor <= 0: plain nearest centroid)
 int stream_kmeans(const Dims& d, int dtype, const void* X, int problems, int C, int kind, uint64_t seed, float beta,
                   int first_batch, int n_batches, float* totals, float* counts, float* centres, int32_t* assign_stream,
-                  cudaStream_t st);
+                  int32_t* status, cudaStream_t st);
 int balanced_assign(const Dims& d, int dtype, const void* X, int problems, int C, int kind, const float* centres, float factor,
                     int32_t* assign, void* ws, cudaStream_t st);
 size_t balanced_ws_bytes(const Dims& d, int problems, int C);

@@ -12,7 +12,7 @@ import torch
 
 from oracle import muse_oracle as orc
 from paper_2509_10406_b200 import workloads as wl
-from tests.gpu_util import Case, to_dev, to_np, tol, rel_err
+from tests.gpu_util import Case, to_dev, to_np, tol, rel_err, kernels_launched
 from tests.test_gpu_cluster import CASES
 
 pytestmark = pytest.mark.gpu
@@ -27,10 +27,20 @@ def _ws(mb, p):
     return torch.zeros(mb.muse_stream_workspace_bytes(p), dtype=torch.uint8, device="cuda")
 
 
-@pytest.mark.parametrize("name", ["tiny", "gqa_bf16", "d128"])
+# shapes that exercise the tensor-core kernel's splits: (centroids per CTA, tiles per CTA) = (128, 1) over 4 CTAs, (256, 2) over
+# 2 CTAs, and ragged slices of 100 centroids over 2 CTAs
+STREAM_CASES = dict(CASES)
+STREAM_CASES.update({
+    "tc_split4": wl.WORKLOADS["headline"].with_(name="s4", B=1, Hq=1, Hkv=1, N=1024, Cq=512, Ck=512, m=4, components=64),
+    "tc_two_tiles": wl.WORKLOADS["small"].with_(name="s2", B=5, Hq=8, Hkv=8, N=1024, Cq=512, Ck=512, m=4, components=64),
+    "tc_ragged": wl.WORKLOADS["headline"].with_(name="sr", B=1, Hq=2, Hkv=2, N=1000, Cq=200, Ck=200, m=4, S=4, components=64),
+})
+
+
+@pytest.mark.parametrize("name", ["tiny", "gqa_bf16", "d128", "tc_split4", "tc_two_tiles", "tc_ragged"])
 def test_streaming_minibatch_teacher_forced(name):
     mb = _mb()
-    c = Case(CASES[name], gain=1.0, cluster=False)
+    c = Case(STREAM_CASES[name], gain=1.0, cluster=False)
     w = c.w
     p = c.params(seed=w.seed)
     ws = _ws(mb, p)
@@ -49,7 +59,9 @@ def test_streaming_minibatch_teacher_forced(name):
                 exp.append(orc.streaming_kmeans(Xf[pr], C, orders[pr], inits[pr], first_batch=s, n_batches=1, totals=t0[pr], counts=c0[pr]))
             tot = to_dev(t0.astype(np.float32), "f32"); cnt = to_dev(c0.astype(np.float32), "f32")
             cen = torch.zeros(P, C, w.D, device="cuda"); a_s = torch.full((P, w.N), -7, dtype=torch.int32, device="cuda")
-            mb.muse_stream_kmeans(p, Xd, side, tot, cnt, cen, ws, beta=0.9, first_batch=s, n_batches=1, assign_stream=a_s)
+            with kernels_launched() as rec:
+                mb.muse_stream_kmeans(p, Xd, side, tot, cnt, cen, ws, beta=0.9, first_batch=s, n_batches=1, assign_stream=a_s)
+            assert rec.names == ({"k_stream_kmeans"} if w.dtype == "f32" else {"k_stream_kmeans_tc"}), rec.names
             torch.cuda.synchronize()
             assert mb.muse_status(ws) == 0
             a_gpu, t_gpu, c_gpu, cen_gpu = to_np(a_s), to_np(tot), to_np(cnt), to_np(cen)
