@@ -84,3 +84,27 @@ def test_head_map(mb):
     p = mb.make_params(B=1, Hq=3, Hkv=2, N=1024, D=64, Cq=8, Ck=16, m=4, head_map=[0, 1, 2])
     out = (ctypes.c_size_t * 6)()
     assert mb.lib().muse_workspace_bytes(ctypes.byref(p), out) == -1
+
+
+def test_streaming_clustering_entry_points_check_their_arguments(mb):
+    p = mb.make_params(B=1, Hq=2, Hkv=1, N=1024, D=64, Cq=8, Ck=16, m=4)
+    L = mb.lib()
+    z, fake, odd = ctypes.c_void_p(0), ctypes.c_void_p(4096), ctypes.c_void_p(4100)
+    need = mb.muse_stream_workspace_bytes(p)
+    assert need % 256 == 0 and need > mb.muse_workspace_bytes(p)[0]          # the balanced step adds its sort and rank arrays
+    assert L.muse_stream_workspace_bytes(ctypes.byref(p), None) == -1
+    # muse_stream_kmeans: side in {0, 1}, beta in (0, 1], pointers present and aligned
+    args = lambda **kw: [kw.get("X", fake), kw.get("side", 0), ctypes.c_float(kw.get("beta", 0.9)), kw.get("first", 0), kw.get("nb", -1),
+                         kw.get("tot", fake), fake, fake, z, kw.get("ws", fake), kw.get("wsb", 1 << 20), z]
+    assert L.muse_stream_kmeans(ctypes.byref(p), *args(side=2)) == -1
+    assert L.muse_stream_kmeans(ctypes.byref(p), *args(beta=0.0)) == -1
+    assert L.muse_stream_kmeans(ctypes.byref(p), *args(beta=1.5)) == -1
+    assert L.muse_stream_kmeans(ctypes.byref(p), *args(X=z)) == -1
+    assert L.muse_stream_kmeans(ctypes.byref(p), *args(tot=odd)) == -1
+    assert L.muse_stream_kmeans(ctypes.byref(p), *args(wsb=16)) == -3
+    # muse_balanced_assign and muse_cluster_streaming: workspace from muse_stream_workspace_bytes
+    assert L.muse_balanced_assign(ctypes.byref(p), fake, 1, fake, ctypes.c_float(4.0), fake, fake, 1024, z) == -3
+    assert L.muse_balanced_assign(ctypes.byref(p), fake, 3, fake, ctypes.c_float(4.0), fake, fake, need, z) == -1
+    assert L.muse_cluster_streaming(ctypes.byref(p), fake, fake, ctypes.c_float(0.9), ctypes.c_float(4.0), fake, fake, fake, fake,
+                                    fake, need - 256, z) == -3
+    assert L.muse_cluster_streaming(ctypes.byref(p), z, z, ctypes.c_float(0.9), ctypes.c_float(4.0), z, z, z, z, fake, need, z) == -1
