@@ -663,6 +663,41 @@ def main():
         context["sharp_inputs_ms_per_step"] = ev0.elapsed_time(ev1) / 3
         context["sharp_inputs_device_status"] = mb.muse_status(buf.ws)
         Q.mul_(1.0 / 128.0)
+    if not args.no_sharp and args.clustering == "lloyd" and args.k2 == 0 and not args.dipole and w.dtype == "bf16" and groups == 1:
+        # the path's two options on the same inputs, device-timed, as context beside the headline numbers: the paper's own
+        # clustering in place of Lloyd (cluster stage only), and the two-level retrieval with k2 = 1 (summarize + forward)
+        try:
+            sws = torch.zeros(mb.muse_stream_workspace_bytes(p), dtype=torch.uint8, device="cuda")
+            for it in range(3):
+                if it == 1:
+                    ev0.record()
+                mb.muse_cluster_streaming(p, Q, K, buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, sws, beta=0.9, cap_factor=4.0)
+            ev1.record(); torch.cuda.synchronize()
+            context["streaming_clustering_stage_ms"] = ev0.elapsed_time(ev1) / 2
+            context["streaming_clustering_device_status"] = mb.muse_status(sws)
+            del sws
+            mb.muse_cluster(p, Q, K, init_q, init_k, buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, buf.ws)
+            p2 = mb.make_params(B=w.B, Hq=hq, Hkv=hkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=w.m, n_blocks=w.S, dtype=w.dtype,
+                                kmeans_iters=w.T, k2=1)
+            need2 = mb.muse_workspace_bytes(p2)
+            if need2[4] < 60e9:
+                aq, ak, qb = buf.assign_q.clone(), buf.assign_k.clone(), buf.qbar.clone()
+                del buf
+                torch.cuda.empty_cache()
+                b2 = mb.MuseBuffers(p2, backward=False)
+                for it in range(3):
+                    if it == 1:
+                        ev0.record()
+                    mb.muse_summarize(p2, K, V, ak, qb, b2.off_k, b2.perm_k, b2.summaries, b2.ws)
+                    mb.muse_attn_fwd(p2, Q, K, V, aq, qb, b2.off_k, b2.perm_k, b2.summaries, None, O_all, b2.LSE, b2.sel, b2.ws,
+                                     bsel_out=b2.bsel)
+                ev1.record(); torch.cuda.synchronize()
+                context["two_level_k2_1_summarize_plus_forward_ms"] = ev0.elapsed_time(ev1) / 2
+                context["k2_all_summarize_plus_forward_ms"] = stages.get("summarize", 0.0) + stages.get("forward", 0.0)
+                context["two_level_device_status"] = mb.muse_status(b2.ws)
+                del b2
+        except Exception as ex:
+            context["options_error"] = repr(ex)[:200]
     context["paper"] = ("2x over cuDNN flash attention at 64k and +36% pretraining throughput, 8xA100, "
                         "D=64, QK128R8SP1B8k (other hardware and configuration: context only)")
 

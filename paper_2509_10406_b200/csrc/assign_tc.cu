@@ -33,7 +33,8 @@ struct AtBars { uint64_t full[4], empty[4], tfull[2], tempty[2], xbar; };
 template <int D>
 __global__ void __launch_bounds__(kAtThreads, 1)
 k_assign_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_hi, const __grid_constant__ CUtensorMap tm_lo,
-            int N, int C, int ns, const float* __restrict__ cnorm, int32_t* __restrict__ assign, int* __restrict__ status) {
+            int N, int C, int ns, const float* __restrict__ cnorm, int32_t* __restrict__ assign, float* __restrict__ dist_out,
+            int* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ AtBars bars;
   __shared__ uint32_t tbase_s;
@@ -116,8 +117,18 @@ k_assign_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
         const int c0 = t * kAtCols + wg * 64 + 32 * q;
 #pragma unroll
         for (int k = 0; k < 32; ++k) {
-          const float dist = fmaf(-2.f, v[k], cn[c0 + k]);
-          if (dist < best) { best = dist; bidx = c0 + k; }     // ascending index: ties keep the lower
+          v[k] = fmaf(-2.f, v[k], cn[c0 + k]);
+          if (v[k] < best) { best = v[k]; bidx = c0 + k; }     // ascending index: ties keep the lower
+        }
+        if (dist_out != nullptr && row0 + row < N) {             // optional output: the whole matrix |c|^2 - 2 x.c
+          float* dr = dist_out + ((size_t)prob * N + row0 + row) * C + c0;
+          if (c0 + 32 <= C && (C & 3) == 0) {
+#pragma unroll
+            for (int k = 0; k < 32; k += 4) *reinterpret_cast<float4*>(dr + k) = make_float4(v[k], v[k + 1], v[k + 2], v[k + 3]);
+          } else {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) if (c0 + k < C) dr[k] = v[k];
+          }
         }
       }
       tc::fence_before_sync();
@@ -143,7 +154,7 @@ k_assign_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
 int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
 
 int assign_tc(const void* X, int problems, int N, int D, int C, const float* centres, const float* cnorm, void* chi,
-              void* clo, int32_t* assign, int* status, cudaStream_t st) {
+              void* clo, int32_t* assign, float* dist_out, int* status, cudaStream_t st) {
   const long long n = (long long)problems * C * D;
   prof_mark("k_split_centres", st);
   k_split_centres<<<(unsigned)((n + 255) / 256), 256, 0, st>>>(centres, n, (bf16*)chi, (bf16*)clo);
@@ -160,10 +171,10 @@ int assign_tc(const void* X, int problems, int N, int D, int C, const float* cen
   prof_mark("k_assign_tc", st);
   if (D == 128) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_assign_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_assign_tc<128><<<grid, kAtThreads, smem, st>>>(tx, thi, tlo, N, C, ns, cnorm, assign, status);
+    k_assign_tc<128><<<grid, kAtThreads, smem, st>>>(tx, thi, tlo, N, C, ns, cnorm, assign, dist_out, status);
   } else {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_assign_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_assign_tc<64><<<grid, kAtThreads, smem, st>>>(tx, thi, tlo, N, C, ns, cnorm, assign, status);
+    k_assign_tc<64><<<grid, kAtThreads, smem, st>>>(tx, thi, tlo, N, C, ns, cnorm, assign, dist_out, status);
   }
   MUSE_LAUNCH_OK();
   return MUSE_OK;

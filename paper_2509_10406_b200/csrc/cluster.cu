@@ -184,7 +184,7 @@ int bucket_sort(int, const int32_t* assign, int problems, int N, int C, int S, i
 // Lloyd iterations
 // ---------------------------------------------------------------------------------------------
 int assign_tc(const void* X, int problems, int N, int D, int C, const float* centres, const float* cnorm, void* chi,
-              void* clo, int32_t* assign, int* status, cudaStream_t st);
+              void* clo, int32_t* assign, float* dist_out, int* status, cudaStream_t st);
 
 template <class T>
 __global__ void k_init_centres(const T* __restrict__ X, int N, int D, int C, const int32_t* __restrict__ init_idx,
@@ -215,7 +215,7 @@ constexpr int kAsgRows = 128, kAsgCols = 64, kAsgThreads = 256;
 template <class T, int D>
 __global__ void __launch_bounds__(kAsgThreads)
 k_assign(const T* __restrict__ X, int N, int C, const float* __restrict__ centres,
-         const float* __restrict__ cnorm, int32_t* __restrict__ assign) {
+         const float* __restrict__ cnorm, int32_t* __restrict__ assign, float* __restrict__ dist_out) {
   constexpr int LD = D + 4;
   extern __shared__ float smf[];
   float* Xs = smf;                       // [128][LD]
@@ -274,6 +274,8 @@ k_assign(const T* __restrict__ X, int N, int C, const float* __restrict__ centre
         float dist = fmaf(-2.f, acc[r][k], cn[tx * 4 + k]);
         int c = c0 + tx * 4 + k;
         if (dist < best[r]) { best[r] = dist; bidx[r] = c; }   // ascending c: ties keep the lower
+        // (optional output: the whole matrix |c|^2 - 2 x.c, for the balanced assignment's second step)
+        if (dist_out != nullptr && c < C && row0 + ty * 8 + r < N) dist_out[((size_t)prob * N + row0 + ty * 8 + r) * C + c] = dist;
       }
   }
 #pragma unroll
@@ -382,7 +384,7 @@ k_update(const T* __restrict__ X, int N, int C, int S, int kind, const int32_t* 
 template <class T, int D>
 static int lloyd_t(const Dims& d, const T* X, int problems, int C, int kind, const int32_t* init_idx,
                    int init_mode, uint64_t seed, int T_iters, int32_t* assign, float* centres, void* ws,
-                   cudaStream_t st) {
+                   float* dist_out, cudaStream_t st) {
   Arena ar(ws);
   int32_t* status = ar.take<int32_t>(kStatusWords);     // cleared by the entry point, shared by both sides
   float* cnorm = ar.take<float>((size_t)problems * C);
@@ -405,11 +407,12 @@ static int lloyd_t(const Dims& d, const T* X, int problems, int C, int kind, con
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_assign<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   for (int it = 0; it <= T_iters; ++it) {
     if (kTensor) {
-      int rc = assign_tc(X, problems, d.N, D, C, centres, cnorm, chi, clo, assign, status, st);
+      int rc = assign_tc(X, problems, d.N, D, C, centres, cnorm, chi, clo, assign, it == T_iters ? dist_out : nullptr, status, st);
       if (rc != MUSE_OK) return rc;
     } else {
       prof_mark("k_assign", st);
-      k_assign<T, D><<<dim3(cdiv(d.N, kAsgRows), problems), kAsgThreads, smem, st>>>(X, d.N, C, centres, cnorm, assign);
+      k_assign<T, D><<<dim3(cdiv(d.N, kAsgRows), problems), kAsgThreads, smem, st>>>(X, d.N, C, centres, cnorm, assign,
+                                                                                          it == T_iters ? dist_out : nullptr);
       MUSE_LAUNCH_OK();
     }
     if (it == T_iters) break;
@@ -435,13 +438,13 @@ size_t lloyd_ws_bytes(const Dims& d, int problems, int C, int) {
 }
 
 int lloyd(const Dims& d, int dtype, const void* X, int problems, int C, int kind, const int32_t* init_idx,
-          int init_mode, uint64_t seed, int T, int32_t* assign, float* centres, void* ws, cudaStream_t st) {
+          int init_mode, uint64_t seed, int T, int32_t* assign, float* centres, void* ws, cudaStream_t st, float* dist_out) {
   if (dtype == MUSE_F32) {
-    if (d.D == 64) return lloyd_t<float, 64>(d, (const float*)X, problems, C, kind, init_idx, init_mode, seed, T, assign, centres, ws, st);
-    return lloyd_t<float, 128>(d, (const float*)X, problems, C, kind, init_idx, init_mode, seed, T, assign, centres, ws, st);
+    if (d.D == 64) return lloyd_t<float, 64>(d, (const float*)X, problems, C, kind, init_idx, init_mode, seed, T, assign, centres, ws, dist_out, st);
+    return lloyd_t<float, 128>(d, (const float*)X, problems, C, kind, init_idx, init_mode, seed, T, assign, centres, ws, dist_out, st);
   }
-  if (d.D == 64) return lloyd_t<__nv_bfloat16, 64>(d, (const __nv_bfloat16*)X, problems, C, kind, init_idx, init_mode, seed, T, assign, centres, ws, st);
-  return lloyd_t<__nv_bfloat16, 128>(d, (const __nv_bfloat16*)X, problems, C, kind, init_idx, init_mode, seed, T, assign, centres, ws, st);
+  if (d.D == 64) return lloyd_t<__nv_bfloat16, 64>(d, (const __nv_bfloat16*)X, problems, C, kind, init_idx, init_mode, seed, T, assign, centres, ws, dist_out, st);
+  return lloyd_t<__nv_bfloat16, 128>(d, (const __nv_bfloat16*)X, problems, C, kind, init_idx, init_mode, seed, T, assign, centres, ws, dist_out, st);
 }
 
 }  // namespace muse

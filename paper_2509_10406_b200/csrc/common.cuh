@@ -148,7 +148,8 @@ int bucket_sort(int dtype_unused, const int32_t* assign, int problems, int N, in
 
 int lloyd(const Dims& d, int dtype, const void* X, int problems, int C, int kind,
           const int32_t* init_idx, int init_mode, uint64_t seed, int T,
-          int32_t* assign, float* centres, void* ws, cudaStream_t st);
+          int32_t* assign, float* centres, void* ws, cudaStream_t st, float* dist_out = nullptr);   // dist_out: [problems, N, C]
+                                                                                               // |c|^2 - 2 x.c of the final assignment (optional)
 size_t lloyd_ws_bytes(const Dims& d, int problems, int C, int kind);
 
 // the paper's own clustering: one streaming pass (state = totals, counts; n_batches < 0: to the end) and the

@@ -16,8 +16,9 @@
 // centroid of every vector (the assignment kernels of the Lloyd path), a stable (block, cluster) counting
 // sort, and each vector's rank inside its bucket in position order; the first cap of a bucket keep it.
 // Step 2: one CTA per (problem, block) walks the displaced vectors in position order and gives each the
-// nearest centroid whose bucket still has room.  Where the cap rarely binds (the paper's regime: 128 clusters,
-// cap 256 per block) step 2 is short; where it binds for most vectors the sequential walk dominates.
+// nearest centroid whose bucket still has room: a masked arg-min over one row of the distance matrix that the
+// step-1 assignment wrote.  Where the cap rarely binds (the paper's regime: 128 clusters, cap 256 per block)
+// step 2 is short; where it binds for most vectors the sequential walk dominates the stage.
 #include <cooperative_groups.h>
 #include "common.cuh"
 #include "feistel.cuh"
@@ -518,29 +519,18 @@ __global__ void k_bucket_rank(const int32_t* __restrict__ assign, const int32_t*
 
 constexpr int kCapThreads = 512;
 
-// x.c_j with the lanes of a warp sharing the D dimensions
-template <int EPL>
-__device__ __forceinline__ float cap_partial(const float (&x)[EPL], const float (&c)[EPL]) {
-  float part = 0.f;
-#pragma unroll
-  for (int k = 0; k < EPL; ++k) part = fmaf(x[k], c[k], part);
-  return part;
-}
-
-template <class T, int D>
+// Step 2: the displaced vectors of one (problem, block), in position order; each takes the nearest centroid whose bucket
+// still has room.  The distances of every vector to every centroid were written by the step-1 assignment, so a placement is
+// a masked arg-min over one row of that matrix (ties to the lower index).
 __global__ void __launch_bounds__(kCapThreads)
-k_cap_overflow(const T* __restrict__ X, int N, int C, int S, int Bs, int cap, const float* __restrict__ centres,
-               const float* __restrict__ cnorm, const int32_t* __restrict__ off, const int32_t* __restrict__ rank,
-               int32_t* __restrict__ assign) {
-  constexpr int EPL = D / 32, NW = kCapThreads / 32;
+k_cap_overflow(int N, int C, int S, int Bs, int cap, const float* __restrict__ dist, const int32_t* __restrict__ off,
+               const int32_t* __restrict__ rank, int32_t* __restrict__ assign) {
+  constexpr int NW = kCapThreads / 32;
   extern __shared__ int cap_smem[];
   int* size = cap_smem;                        // [C] bucket sizes of this block
   __shared__ int lst[kCapThreads], wcnt[NW], ri[NW];
-  __shared__ float xs[D], rd[NW];
+  __shared__ float rd[NW];
   const int b = blockIdx.x, prob = blockIdx.y, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const T* Xp = X + (size_t)prob * N * D;
-  const float* Cp = centres + (size_t)prob * C * D;
-  const float* cn = cnorm + (size_t)prob * C;
   const int32_t* o = off + (size_t)prob * (C * S + 1) + (size_t)b * C;
   const int32_t* rk = rank + (size_t)prob * N;
   int32_t* as = assign + (size_t)prob * N;
@@ -559,39 +549,19 @@ k_cap_overflow(const T* __restrict__ X, int N, int C, int S, int Bs, int cap, co
     __syncthreads();
     for (int e = 0; e < total; ++e) {
       const int u = lst[e];
-      if (tid < D) xs[tid] = to_f(Xp[(size_t)u * D + tid]);
-      __syncthreads();
+      const float* dr = dist + ((size_t)prob * N + u) * C;
       float best = INFINITY;
       int bj = 0x7fffffff;
-      float x[EPL];
+      for (int j = tid; j < C; j += kCapThreads) {
+        if (size[j] >= cap) continue;
+        const float dv = dr[j];
+        if (dv < best) { best = dv; bj = j; }                          // (ascending j per thread)
+      }
 #pragma unroll
-      for (int k = 0; k < EPL; ++k) x[k] = xs[lane * EPL + k];
-      for (int j0 = warp; j0 < C; j0 += 4 * NW) {                      // four centroid rows in flight per warp
-        float c[4][EPL], part[4];
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          const int j = j0 + r * NW;
-          if (j < C && size[j] < cap) ldv<EPL>(Cp + (size_t)j * D + lane * EPL, c[r]);      // (warp-uniform)
-          else {
-#pragma unroll
-            for (int k = 0; k < EPL; ++k) c[r][k] = 0.f;
-          }
-        }
-#pragma unroll
-        for (int r = 0; r < 4; ++r) part[r] = cap_partial<EPL>(x, c[r]);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-          for (int r = 0; r < 4; ++r) part[r] += __shfl_xor_sync(0xffffffffu, part[r], o);
-        }
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-          const int j = j0 + r * NW;
-          if (j < C && size[j] < cap) {
-            const float dist = fmaf(-2.f, part[r], cn[j]);
-            if (dist < best) { best = dist; bj = j; }                  // (ascending j within the warp)
-          }
-        }
+      for (int o2 = 16; o2 > 0; o2 >>= 1) {
+        const float ob = __shfl_xor_sync(0xffffffffu, best, o2);
+        const int oj = __shfl_xor_sync(0xffffffffu, bj, o2);
+        if (ob < best || (ob == best && oj < bj)) { best = ob; bj = oj; }
       }
       if (lane == 0) { rd[warp] = best; ri[warp] = bj; }
       __syncthreads();
@@ -600,7 +570,7 @@ k_cap_overflow(const T* __restrict__ X, int N, int C, int S, int Bs, int cap, co
         int bi = ri[0];
         for (int w = 1; w < NW; ++w)
           if (rd[w] < bd || (rd[w] == bd && ri[w] < bi)) { bd = rd[w]; bi = ri[w]; }
-        if ((unsigned)bi >= (unsigned)C)                             // every distance was NaN: first centroid with room
+        if ((unsigned)bi >= (unsigned)C)                               // every distance was NaN: first centroid with room
           for (bi = 0; bi < C - 1 && size[bi] >= cap; ++bi) {}
         as[u] = bi;
         size[bi] += 1;
@@ -608,15 +578,6 @@ k_cap_overflow(const T* __restrict__ X, int N, int C, int S, int Bs, int cap, co
       __syncthreads();
     }
   }
-}
-
-__global__ void k_centre_norms2(const float* __restrict__ centres, int total, int D, float* __restrict__ cnorm) {
-  const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (w >= total) return;
-  float n2 = 0.f;
-  for (int d = lane; d < D; d += 32) { const float v = centres[(size_t)w * D + d]; n2 = fmaf(v, v, n2); }
-  n2 = warp_sum(n2);
-  if (lane == 0) cnorm[w] = n2;
 }
 
 size_t balanced_ws_bytes(const Dims& d, int problems, int C) {
@@ -627,41 +588,33 @@ size_t balanced_ws_bytes(const Dims& d, int problems, int C) {
   ar.take<int32_t>((size_t)problems * d.N);
   ar.take<int32_t>((size_t)problems * sort_ws_elems(d.N, C * d.S));
   ar.take<int32_t>((size_t)problems * d.N);
+  ar.take<float>((size_t)problems * d.N * C);
   return ar.used;
 }
 
 int balanced_assign(const Dims& d, int dtype, const void* X, int problems, int C, int kind, const float* centres, float factor,
                     int32_t* assign, void* ws, cudaStream_t st) {
-  // step 1a: nearest centroid of every vector (the Lloyd path's final assignment against given centres)
-  int rc = lloyd(d, dtype, X, problems, C, kind, nullptr, MUSE_INIT_CENTRES, 0, 0, assign, const_cast<float*>(centres), ws, st);
-  if (rc != MUSE_OK || !(factor > 0.f)) return rc;
-  const int cap = (int)ceil((double)factor * d.Bs / C);
-  if (cap >= d.Bs) return MUSE_OK;             // the cap cannot bind
+  const int cap = factor > 0.f ? (int)ceil((double)factor * d.Bs / C) : d.Bs;
+  const bool binds = cap < d.Bs;               // otherwise the cap cannot bind: plain nearest centroid
   Arena ar(ws);
   ar.take<char>(lloyd_ws_bytes(d, problems, C, 0));
-  float* cnorm = ar.take<float>((size_t)problems * C);
+  ar.take<float>((size_t)problems * C);
   int32_t* off = ar.take<int32_t>((size_t)problems * (C * d.S + 1));
   int32_t* perm = ar.take<int32_t>((size_t)problems * d.N);
   int32_t* scratch = ar.take<int32_t>((size_t)problems * sort_ws_elems(d.N, C * d.S));
   int32_t* rank = ar.take<int32_t>((size_t)problems * d.N);
+  float* dist = ar.take<float>((size_t)problems * d.N * C);      // |c|^2 - 2 x.c of every (vector, centroid), written by step 1
+  // step 1a: nearest centroid of every vector (the Lloyd path's final assignment against given centres)
+  int rc = lloyd(d, dtype, X, problems, C, kind, nullptr, MUSE_INIT_CENTRES, 0, 0, assign, const_cast<float*>(centres), ws, st,
+                 binds ? dist : nullptr);
+  if (rc != MUSE_OK || !binds) return rc;
   rc = bucket_sort(0, assign, problems, d.N, C, d.S, d.Bs, 0, off, perm, scratch, st);      // key = block * C + cluster
   if (rc != MUSE_OK) return rc;
   prof_mark("k_bucket_rank", st);
   k_bucket_rank<<<dim3(cdiv(d.N, 256), problems), 256, 0, st>>>(assign, off, perm, d.N, C, d.S, d.Bs, rank);
   MUSE_LAUNCH_OK();
-  k_centre_norms2<<<cdiv(problems * C * 32, 256), 256, 0, st>>>(centres, problems * C, d.D, cnorm);
-  MUSE_LAUNCH_OK();
-  const size_t smem = (size_t)C * sizeof(int);
-  typedef __nv_bfloat16 bf;
-  const dim3 grid(d.S, problems);
   prof_mark("k_cap_overflow", st);
-  if (dtype == MUSE_F32) {
-    if (d.D == 64) k_cap_overflow<float, 64><<<grid, kCapThreads, smem, st>>>((const float*)X, d.N, C, d.S, d.Bs, cap, centres, cnorm, off, rank, assign);
-    else k_cap_overflow<float, 128><<<grid, kCapThreads, smem, st>>>((const float*)X, d.N, C, d.S, d.Bs, cap, centres, cnorm, off, rank, assign);
-  } else {
-    if (d.D == 64) k_cap_overflow<bf, 64><<<grid, kCapThreads, smem, st>>>((const bf*)X, d.N, C, d.S, d.Bs, cap, centres, cnorm, off, rank, assign);
-    else k_cap_overflow<bf, 128><<<grid, kCapThreads, smem, st>>>((const bf*)X, d.N, C, d.S, d.Bs, cap, centres, cnorm, off, rank, assign);
-  }
+  k_cap_overflow<<<dim3(d.S, problems), kCapThreads, (size_t)C * sizeof(int), st>>>(d.N, C, d.S, d.Bs, cap, dist, off, rank, assign);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }
