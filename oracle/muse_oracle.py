@@ -22,7 +22,8 @@ Readings taken where the paper is silent (listed again in the design notes):
  * spatial selection k_2 = all causally visible blocks on the hot path, so the merge has three
    non-empty components (far approximation, retrieved exact, local exact).  forward(k2 > 0)
    also states the two-level retrieval (block selection with per-block summaries and the
-   fourth, near-field component); block ties go to the lower block index.  Forward only.
+   fourth, near-field component); block ties go to the lower block index.  backward(k2 > 0)
+   holds the chosen blocks constant like the chosen clusters.
  * top-m: among clusters with at least one visible key, largest score first,
    ties to the lower cluster index; fewer than m candidates -> take them all.
 
@@ -34,7 +35,9 @@ test); key-translation invariance; weights sum to one and are causal;
 error bilinear in the residuals; backward vs central finite differences and,
 for m = C_k, vs the closed-form dense-attention gradient.  Two-level retrieval: k2 >= S - 1
 reproduces k2 = all; a separately written single softmax over exact and stand-in keys on tiny
-inputs; singleton key or query clusters stay exact for every k2; weights causal, sum to one.  Dipole: the Jacobian
+inputs; singleton key or query clusters stay exact for every k2; weights causal, sum to one; its
+backward vs central finite differences with clusters and blocks held fixed, and k2 >= S - 1 vs the
+single-level backward.  Dipole: the Jacobian
 of the far field at zero residual equals the dense-attention Jacobian (a
 cross-covariance written separately in the test), the error falls from first
 to second order in the residual, causality and key-translation invariance.  Streaming k-means: closed-form
@@ -431,12 +434,14 @@ def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs
     ret_mask = vis[None, :] & selmask[:, a_k]
     o_near = np.zeros((len(rows), V.shape[1])); lse_near = np.full(len(rows), -np.inf)
     bsel = None
+    near_logit = None
     if k2 > 0 and causal:
         # 2. block selection inside the selected clusters, with the pre-accumulation summaries
         mu_b, ka_b, nu_b = blk_i                           # [S, Ck], [S, Ck, D], [S, Ck, Dv]
         bsel = np.full((len(rows), max(m, 1), k2), -1, np.int32)
         blk_of = u // Bs
         ret_mask = np.zeros((len(rows), N), bool)
+        near_logit = np.full((len(rows), max(b, 1), Ck), -np.inf)   # logit of the stand-in key (b', j) for each query
         for r in range(len(rows)):
             near_logits, near_values = [], []
             for k, j in enumerate(sel_rows[r]):
@@ -455,6 +460,7 @@ def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs
                         ret_mask[r] |= (a_k == j) & (blk_of == bp)
                     else:                                  # not retrieved: its per-block summary stands in
                         near_logits.append(bl[bp]); near_values.append(nu_b[bp, j])
+                        near_logit[r, bp, j] = bl[bp]
             if near_logits:
                 o1, l1 = _softmax_part(np.asarray(near_logits)[None, :], np.asarray(near_values))
                 o_near[r], lse_near[r] = o1[0], l1[0]
@@ -473,7 +479,7 @@ def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs
     L = _lse(lses, 1)
     wts = np.exp(lses - L[:, None])
     O = wts[:, 0:1] * o_far + wts[:, 1:2] * o_ret + wts[:, 2:3] * o_loc + wts[:, 3:4] * o_near
-    return dict(O=O, L=L, sel=sel_rows, bsel=bsel, o_near=o_near, lse_near=lse_near, sel_gap=gap, selmask=selmask, score=score, qp=qp, qres=qres,
+    return dict(O=O, L=L, sel=sel_rows, bsel=bsel, near_logit=near_logit, o_near=o_near, lse_near=lse_near, sel_gap=gap, selmask=selmask, score=score, qp=qp, qres=qres,
                 far_logit=far_logit, exact_logit=np.where(ret_mask | loc_mask, logit, -np.inf),
                 o_far=o_far, lse_far=lse_far, o_ret=o_ret, lse_ret=lse_ret,
                 o_loc=o_loc, lse_loc=lse_loc)
@@ -543,11 +549,13 @@ def forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, 
 
 
 def backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, sel_mode=0,
-             agg_grad=True, rows=None):
+             agg_grad=True, rows=None, k2=0, bsel=None):
     """Gradients of sum(O * dO) w.r.t. Q, K, V with the assignments, the selections and the
     query centroids held constant (Appendix "Centroid Gradient Flow"; assignments and
     selections are discrete).  agg_grad=False also treats the tilted aggregation weights as
-    constants (Appendix "Aggregation Weight Gradient Flow").  Returns (dQ, dK, dV, fwd)."""
+    constants (Appendix "Aggregation Weight Gradient Flow").  k2 > 0: two-level retrieval; the
+    chosen blocks (`bsel`) are constants like the clusters, and the stand-in keys of the other
+    blocks pass their gradient on through the per-block summaries.  Returns (dQ, dK, dV, fwd)."""
     Q = np.asarray(Q, np.float64); K = np.asarray(K, np.float64); V = np.asarray(V, np.float64)
     dO = np.asarray(dO, np.float64); qbar = np.asarray(qbar, np.float64)
     N, D = Q.shape; Dv = V.shape[1]; Cq = qbar.shape[0]
@@ -555,6 +563,10 @@ def backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=N
         S = 1
     Bs = N // S
     muh, kah, nuh = accumulated_summaries(K, V, a_k, qbar, sigma, S, Ck, causal)
+    two_level = k2 > 0 and causal
+    if two_level:
+        mu_b, ka_b, nu_b = block_summaries(K, V, a_k, qbar, sigma, S, Ck)
+        dmu_b = np.zeros_like(mu_b); dka_b = np.zeros_like(ka_b); dnu_b = np.zeros_like(nu_b)
     dQ = np.zeros((N, D)); dK = np.zeros((N, D)); dV = np.zeros((N, Dv))
     dmu = np.zeros_like(muh); dka = np.zeros_like(kah); dnu = np.zeros_like(nuh)
     fwd = dict(O=np.zeros((N, Dv)), LSE=np.full(N, -np.inf), sel=np.full((N, m), -1, np.int32),
@@ -562,7 +574,9 @@ def backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=N
     for b, i, r in _segments(a_q, N, S, causal, rows):
         seg = _segment(Q, K, V, a_k, qbar[i], muh[b, i], kah[b, i], nuh[b, i], r, b,
                        sigma=sigma, Bs=Bs, m=m, causal=causal,
-                       sel_rows=None if sel is None else sel[r], sel_mode=sel_mode)
+                       sel_rows=None if sel is None else sel[r], sel_mode=sel_mode, k2=k2 if two_level else 0,
+                       blk_i=(mu_b[:, i], ka_b[:, i], nu_b[:, i]) if two_level else None,
+                       bsel_rows=None if bsel is None else bsel[r])
         fwd["O"][r], fwd["LSE"][r], fwd["sel"][r] = seg["O"], seg["L"], seg["sel"]
         fwd["sel_gap"][r] = seg["sel_gap"]
         L = seg["L"][:, None]
@@ -580,6 +594,16 @@ def backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=N
         dqp += Gf @ kah[b, i]                              # d score / d q = kah (qbar constant)
         dka[b, i] += Gf.T @ seg["qres"]
         dmu[b, i] += Gf.sum(0)
+        if two_level and seg["near_logit"] is not None:
+            # the stand-in keys (b', j) of the non-retrieved blocks of the selected clusters: logit
+            # qres . kappa_b'j + mu_b'j, value nu_b'j (per-block summaries of this query cluster)
+            for bp in range(b):
+                Pn = np.exp(seg["near_logit"][:, bp, :] - L)       # [n, Ck], zero where there is no stand-in key
+                dnu_b[bp, i] += Pn.T @ g_out
+                Gn = Pn * (g_out @ nu_b[bp, i].T - delta)
+                dqp += Gn @ ka_b[bp, i]
+                dka_b[bp, i] += Gn.T @ seg["qres"]
+                dmu_b[bp, i] += Gn.sum(0)
         dQ[r] = sigma * dqp
     # through the accumulated summaries to the keys and values they were built from
     blk = np.arange(N) // Bs
@@ -598,6 +622,22 @@ def backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=N
                           + dka[b, :, j] @ K[mem].T - (dka[b, :, j] * kah[b, :, j]).sum(1)[:, None]
                           + dnu[b, :, j] @ V[mem].T - (dnu[b, :, j] * nuh[b, :, j]).sum(1)[:, None])
                 dK[mem] += sigma * (dl.T @ qbar)
+    if two_level:
+        # ... and through the per-block summaries to the keys and values of their own bucket
+        for bp in range(S):
+            for j in range(Ck):
+                mem = np.nonzero((blk == bp) & (a_k == j))[0]
+                if mem.size == 0:
+                    continue
+                l = sigma * (qbar @ K[mem].T)
+                w = np.exp(l - mu_b[bp, :, j][:, None])
+                dK[mem] += w.T @ dka_b[bp, :, j]
+                dV[mem] += w.T @ dnu_b[bp, :, j]
+                if agg_grad:
+                    dl = w * (dmu_b[bp, :, j][:, None]
+                              + dka_b[bp, :, j] @ K[mem].T - (dka_b[bp, :, j] * ka_b[bp, :, j]).sum(1)[:, None]
+                              + dnu_b[bp, :, j] @ V[mem].T - (dnu_b[bp, :, j] * nu_b[bp, :, j]).sum(1)[:, None])
+                    dK[mem] += sigma * (dl.T @ qbar)
     return dQ, dK, dV, fwd
 
 
@@ -627,7 +667,7 @@ def layer_forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=
 
 
 def layer_backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None,
-                   sel_mode=0, agg_grad=True, head_map=None):
+                   sel_mode=0, agg_grad=True, head_map=None, k2=0, bsel=None):
     """dK, dV of a kv head are the sums over the query heads that share it."""
     B, Hq, N, D = Q.shape
     Hkv = K.shape[1]
@@ -639,7 +679,7 @@ def layer_backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True,
             q, k, v, _ = backward(Q[b, h], K[b, g], V[b, g], dO[b, h], a_q[b, h], a_k[b, g],
                                   qbar[b, h], sigma=sigma, S=S, Ck=Ck, m=m, causal=causal,
                                   sel=None if sel is None else sel[b, h], sel_mode=sel_mode,
-                                  agg_grad=agg_grad)
+                                  agg_grad=agg_grad, k2=k2, bsel=None if bsel is None else bsel[b, h])
             dQ[b, h] = q
             dK[b, g] += k
             dV[b, g] += v

@@ -150,3 +150,63 @@ def test_two_level_argument_rules():
         orc.forward(p["Q"], p["K"], p["V"], p["a_q"], p["a_k"], p["qbar"], sigma=p["sigma"], S=p["S"], Ck=p["Ck"], m=2, k2=-1)
     with pytest.raises(ValueError):
         orc.forward(p["Q"], p["K"], p["V"], p["a_q"], p["a_k"], p["qbar"], sigma=p["sigma"], S=p["S"], Ck=p["Ck"], m=0, k2=1, dipole=1)
+
+
+# ------------------------------------------------------------------ backward with two-level retrieval
+
+def _fd(fun, X, h=1e-5):
+    import itertools
+    g = np.zeros_like(X)
+    for idx in itertools.product(*map(range, X.shape)):
+        old = X[idx]
+        X[idx] = old + h; fp = fun()
+        X[idx] = old - h; fm = fun()
+        X[idx] = old
+        g[idx] = (fp - fm) / (2 * h)
+    return g
+
+
+@pytest.mark.parametrize("m,k2,agg", [(2, 1, True), (3, 2, True), (2, 1, False)])
+def test_two_level_backward_matches_finite_differences(m, k2, agg):
+    """Central differences of sum(O * dO) with the chosen clusters and blocks held fixed.  With agg = False the
+    reference forward rebuilds both kinds of summaries with the tilt weights frozen at their initial values."""
+    p = toy_problem(23, N=40, D=4, Dv=3, Cq=3, Ck=4, S=5, gain=2.0)
+    N, S, Ck, sg = p["N"], p["S"], p["Ck"], p["sigma"]
+    kw = dict(sigma=sg, S=S, Ck=Ck, m=m, k2=k2)
+    f0 = orc.forward(p["Q"], p["K"], p["V"], p["a_q"], p["a_k"], p["qbar"], **kw)
+    sel, bsel = f0["sel"], f0["bsel"]
+    assert (bsel >= 0).any() and np.isfinite(f0["lse_near"]).any()          # both kinds of key occur
+    Q, K, V = p["Q"].copy(), p["K"].copy(), p["V"].copy()
+    K0 = p["K"].copy()
+    Bs = N // S
+    blk = np.arange(N) // Bs
+
+    def frozen(kind):
+        """accumulated ('acc') or per-block ('blk') summaries with weights from K0 and the original log-masses"""
+        mu0 = f0["summ"][0] if kind == "acc" else orc.block_summaries(K0, p["V"], p["a_k"], p["qbar"], sg, S, Ck)[0]
+        ka = np.zeros((S, p["Cq"], Ck, p["D"])); nu = np.zeros((S, p["Cq"], Ck, V.shape[1]))
+        for b in range(S):
+            for j in range(Ck):
+                mem = np.nonzero(((blk < b) if kind == "acc" else (blk == b)) & (p["a_k"] == j))[0]
+                if mem.size:
+                    w = np.exp(sg * p["qbar"] @ K0[mem].T - mu0[b, :, j][:, None])
+                    ka[b, :, j] = w @ K[mem]; nu[b, :, j] = w @ V[mem]
+        return mu0, ka, nu
+
+    def loss():
+        extra = {} if agg else dict(summ=frozen("acc"), blocks=frozen("blk"))
+        return (orc.forward(Q, K, V, p["a_q"], p["a_k"], p["qbar"], sel=sel, bsel=bsel, **extra, **kw)["O"] * p["dO"]).sum()
+    dQ, dK, dV, fwd = orc.backward(Q, K, V, p["dO"], p["a_q"], p["a_k"], p["qbar"], sel=sel, bsel=bsel, agg_grad=agg, **kw)
+    np.testing.assert_allclose(fwd["O"], f0["O"], atol=1e-13)
+    for g, X in ((dQ, Q), (dK, K), (dV, V)):
+        fd = _fd(loss, X)
+        assert np.abs(g - fd).max() <= 1e-6 * np.abs(fd).max()
+
+
+def test_two_level_backward_with_every_block_chosen_is_the_single_level_backward():
+    p = toy_problem(24, N=32, D=4, Dv=3, Cq=3, Ck=4, S=4, gain=2.0)
+    kw = dict(sigma=p["sigma"], S=p["S"], Ck=p["Ck"], m=2)
+    a = orc.backward(p["Q"], p["K"], p["V"], p["dO"], p["a_q"], p["a_k"], p["qbar"], **kw)
+    b = orc.backward(p["Q"], p["K"], p["V"], p["dO"], p["a_q"], p["a_k"], p["qbar"], k2=p["S"] - 1, **kw)
+    for x, y in zip(a[:3], b[:3]):
+        np.testing.assert_allclose(x, y, atol=1e-12)
