@@ -296,7 +296,7 @@ def main():
                          "(0 = as few as keep the summaries under 64 GB)")
     ap.add_argument("--forward-only", action="store_true", help="time cluster + summarize + forward only")
     ap.add_argument("--k2", type=int, default=0,
-                    help="spatial blocks retrieved inside each selected cluster (0 = all; > 0 is forward only)")
+                    help="spatial blocks retrieved inside each selected cluster (0 = all visible blocks)")
     ap.add_argument("--clustering", default="lloyd", choices=["lloyd", "streaming"],
                     help="lloyd = muse_cluster (the measured path); streaming = the paper's one-pass mini-batch k-means "
                          "with the balanced per-block assignment (muse_cluster_streaming; device-timed line only)")
@@ -315,8 +315,6 @@ def main():
         w = w.with_(m=args.m)
     if args.dipole:
         w = w.with_(m=0)
-        args.forward_only = True
-    if args.k2 > 0:
         args.forward_only = True
     if args.clustering == "streaming":                    # a device-timed comparison line: no staged run, no oracle sample
         args.no_e2e = True
@@ -391,7 +389,7 @@ def main():
             m_("forward")
             if not args.forward_only:
                 mb.muse_attn_bwd(p, Qg, Kg, Vg, O_all[:, qs], buf.LSE, dO[:, qs], buf.assign_q, buf.qbar, buf.off_k,
-                                 buf.perm_k, buf.summaries, buf.sel, dQ_all[:, qs], dK_all[:, ks], dV_all[:, ks], buf.ws)
+                                 buf.perm_k, buf.summaries, buf.sel, dQ_all[:, qs], dK_all[:, ks], dV_all[:, ks], buf.ws, bsel=buf.bsel)
                 m_("backward")
 
     def barrier():
@@ -503,7 +501,7 @@ def main():
                 if not args.forward_only:
                     cur.wait_event(e_do)
                     mb.muse_attn_bwd(ep, Qg, Kg, Vg, O_all[:, qs], ebuf.LSE, dO[:, qs], ebuf.assign_q, ebuf.qbar, ebuf.off_k,
-                                     ebuf.perm_k, ebuf.summaries, ebuf.sel, dQ_all[:, qs], dK_all[:, ks], dV_all[:, ks], ebuf.ws)
+                                     ebuf.perm_k, ebuf.summaries, ebuf.sel, dQ_all[:, qs], dK_all[:, ks], dV_all[:, ks], ebuf.ws, bsel=ebuf.bsel)
                     e_g = torch.cuda.Event(); e_g.record(cur)
                     with torch.cuda.stream(s_out):
                         s_out.wait_event(e_g)

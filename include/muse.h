@@ -213,9 +213,12 @@ MUSE_API int muse_attn_fwd(const muse_params_t* p, const void* Q, const void* K,
                   const int32_t* sel_in, const int32_t* bsel_in, void* O, float* LSE, int32_t* sel_out,
                   int32_t* bsel_out, void* ws, size_t ws_bytes, cudaStream_t stream);
 
-/* Backward of sum(O * dO) w.r.t. Q, K, V with assign_*, sel and qbar constant; dK, dV of a
+/* Backward of sum(O * dO) w.r.t. Q, K, V with assign_*, sel, bsel and qbar constant; dK, dV of a
  * kv head are summed over the query heads that share it.
  *   O, LSE, sel  in   as returned by muse_attn_fwd (sel must be the selection used there)
+ *   bsel         in   k2 > 0: the chosen blocks [B,Hq,N,m,k2] as returned by muse_attn_fwd (required);
+ *                     ignored (may be NULL) when k2 == 0.  With k2 > 0 the stand-in keys of the
+ *                     non-retrieved blocks pass their gradient on through the per-block summaries
  *   summaries    in   as written by muse_summarize, or NULL: the summaries are then rebuilt from
  *                     K, V, off_k, perm_k, qbar inside the scratch, which must hold
  *                     muse_workspace_bytes out[5] bytes instead of out[3]
@@ -224,7 +227,7 @@ MUSE_API int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K,
                   const void* O, const float* LSE, const void* dO,
                   const int32_t* assign_q, const float* qbar,
                   const int32_t* off_k, const int32_t* perm_k, const void* summaries,
-                  const int32_t* sel, void* dQ, void* dK, void* dV,
+                  const int32_t* sel, const int32_t* bsel, void* dQ, void* dK, void* dV,
                   void* ws, size_t ws_bytes, cudaStream_t stream);
 
 /* The paper's own clustering (Appendix "Clustering Details").  An alternative to muse_cluster with the

@@ -89,7 +89,7 @@ def lib() -> ctypes.CDLL:
         L.muse_cluster.argtypes = [pp, vp, vp, i32p, i32p, i32p, i32p, f32p, f32p, vp, sz, vp]
         L.muse_summarize.argtypes = [pp, vp, vp, i32p, f32p, i32p, i32p, i32p, f32p, f32p, vp, vp, sz, vp]
         L.muse_attn_fwd.argtypes = [pp, vp, vp, vp, i32p, f32p, i32p, i32p, vp, i32p, i32p, vp, f32p, i32p, i32p, vp, sz, vp]
-        L.muse_attn_bwd.argtypes = [pp, vp, vp, vp, vp, f32p, vp, i32p, f32p, i32p, i32p, vp, i32p, vp, vp, vp,
+        L.muse_attn_bwd.argtypes = [pp, vp, vp, vp, vp, f32p, vp, i32p, f32p, i32p, i32p, vp, i32p, i32p, vp, vp, vp,
                                     vp, sz, vp]
         fl, ci = ctypes.c_float, ctypes.c_int
         L.muse_stream_workspace_bytes.argtypes = [pp, ctypes.POINTER(sz)]
@@ -248,9 +248,9 @@ def muse_attn_fwd(p, Q, K, V, assign_q, qbar, off_k, perm_k, summaries, sel_in, 
                                _ptr(bsel_out), _ptr(ws), ws.numel() * ws.element_size(), _stream()), "muse_attn_fwd")
 
 
-def muse_attn_bwd(p, Q, K, V, O, LSE, dO, assign_q, qbar, off_k, perm_k, summaries, sel, dQ, dK, dV, ws):
+def muse_attn_bwd(p, Q, K, V, O, LSE, dO, assign_q, qbar, off_k, perm_k, summaries, sel, dQ, dK, dV, ws, bsel=None):
     _check(lib().muse_attn_bwd(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(O), _ptr(LSE), _ptr(dO),
-                               _ptr(assign_q), _ptr(qbar), _ptr(off_k), _ptr(perm_k), _ptr(summaries), _ptr(sel),
+                               _ptr(assign_q), _ptr(qbar), _ptr(off_k), _ptr(perm_k), _ptr(summaries), _ptr(sel), _ptr(bsel),
                                _ptr(dQ), _ptr(dK), _ptr(dV), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
            "muse_attn_bwd")
 
@@ -310,5 +310,5 @@ def muse_layer_forward(p, buf: MuseBuffers, Q, K, V, init_q=None, init_k=None, s
 
 def muse_layer_backward(p, buf: MuseBuffers, Q, K, V, dO, sel=None):
     muse_attn_bwd(p, Q, K, V, buf.O, buf.LSE, dO, buf.assign_q, buf.qbar, buf.off_k, buf.perm_k, buf.summaries,
-                  buf.sel if sel is None else sel, buf.dQ, buf.dK, buf.dV, buf.ws)
+                  buf.sel if sel is None else sel, buf.dQ, buf.dK, buf.dV, buf.ws, bsel=buf.bsel)
     return buf.dQ, buf.dK, buf.dV

@@ -308,14 +308,14 @@ int muse_attn_fwd(const muse_params_t* p, const void* Q, const void* K, const vo
 int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K, const void* V, const void* O,
                   const float* LSE, const void* dO, const int32_t* assign_q, const float* qbar,
                   const int32_t* off_k, const int32_t* perm_k, const void* summaries, const int32_t* sel,
-                  void* dQ, void* dK, void* dV, void* ws, size_t ws_bytes, cudaStream_t stream) {
+                  const int32_t* bsel, void* dQ, void* dK, void* dV, void* ws, size_t ws_bytes, cudaStream_t stream) {
   Dims d;
   int rc = resolve(p, &d);
   if (rc != MUSE_OK) return rc;
   if (!Q || !K || !V || !O || !LSE || !dO || !assign_q || !qbar || !off_k || !perm_k || !dQ || !dK || !dV || !ws) return MUSE_ERR_INVALID_ARG;
   if (d.dipole) return MUSE_ERR_UNSUPPORTED;       // no backward through the dipole correction
-  if (d.k2 > 0) return MUSE_ERR_UNSUPPORTED;       // nor, yet, through the spatial block selection (forward only)
   if (d.m > 0 && d.SB > 0 && sel == nullptr) return MUSE_ERR_INVALID_ARG;
+  if (d.k2 > 0 && d.m > 0 && d.SB > 0 && bsel == nullptr) return MUSE_ERR_INVALID_ARG;   // the forward pass's chosen blocks
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(qbar) ||
       !aligned16(summaries) || !aligned16(dQ) || !aligned16(dK) || !aligned16(dV) || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;
   size_t need[6];
@@ -331,7 +331,7 @@ int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K, const vo
     if (rc != MUSE_OK) return rc;
     summaries = tail;
   }
-  rc = attn_bwd(d, p->dtype, Q, K, V, O, LSE, dO, assign_q, qbar, off_k, perm_k, summaries, sel, dQ, dK, dV, ws, stream);
+  rc = attn_bwd(d, p->dtype, Q, K, V, O, LSE, dO, assign_q, qbar, off_k, perm_k, summaries, sel, bsel, dQ, dK, dV, ws, stream);
   prof_mark(nullptr, stream);
   return rc;
 }

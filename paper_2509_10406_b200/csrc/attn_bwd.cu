@@ -8,6 +8,10 @@
 
 namespace muse {
 
+int near_bwd(const Dims& d, int dtype, const void* Q, const void* dO, const float* qbar, const float* LSE, const float* delta,
+             const int32_t* off_q, const int32_t* perm_q, const int32_t* sel, const int32_t* bsel, const SummPtrs& sp, float* dQacc,
+             float* dkappa_b, float* dnu_b, float* dS_b, cudaStream_t st);
+
 __device__ __forceinline__ int query_plane_b(const Dims& d, int t) { return d.causal ? t / d.Bs - 1 : 0; }
 
 template <int D>
@@ -465,7 +469,9 @@ __global__ void __launch_bounds__(kFlashThreads)
 k_summ_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const int32_t* __restrict__ off_k,
            const int32_t* __restrict__ off_q, const float* __restrict__ qbar, const float* __restrict__ mu,
            const GT* __restrict__ dkappa, const GT* __restrict__ dnu, const float* __restrict__ dS,
-           float* __restrict__ dK_perm, float* __restrict__ dV_perm) {
+           float* __restrict__ dK_perm, float* __restrict__ dV_perm, int per_block) {
+  // per_block = 1: mu and the gradients belong to the PER-BLOCK summaries (two-level retrieval): bucket b' feeds only
+  // its own summary, so there is no suffix over the planes (the factor below is zero)
   constexpr int LD = D + 4;
   extern __shared__ __align__(16) unsigned char smraw[];
   float* qb = (float*)smraw; float* GU = qb + kTile * LD; float* GW = GU + kTile * LD;
@@ -499,12 +505,13 @@ k_summ_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const in
         float f = 0.f; int lv = 0; float m_here = -INFINITY;
         if (i < dm.Cq) {
           m_here = mu[(((size_t)pq * dm.SB + pl) * dm.Cq + i) * dm.Ck + j];
-          f = (m_here == -INFINITY || muref[tid] == INFINITY) ? 0.f : expf(m_here - muref[tid]);
+          f = (per_block || m_here == -INFINITY || muref[tid] == INFINITY) ? 0.f : expf(m_here - muref[tid]);
           const int blk = dm.causal ? pl + 1 : 0;
-          lv = oq[(size_t)blk * dm.Cq + i + 1] > oq[(size_t)blk * dm.Cq + i] && m_here != -INFINITY;
+          lv = (per_block || oq[(size_t)blk * dm.Cq + i + 1] > oq[(size_t)blk * dm.Cq + i]) && m_here != -INFINITY;
         }
         fac[tid] = f; live[tid] = lv;
         if (m_here != -INFINITY) muref[tid] = m_here;
+        else if (per_block) muref[tid] = INFINITY;       // an empty bucket has no weights of its own
       }
       __syncthreads();
       for (int e = tid; e < kTile * (D / 4); e += kFlashThreads) {
@@ -586,7 +593,7 @@ k_summ_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const in
 // ---------------------------------------------------------------------------------------------
 template <class T, int D, class PT>      // PT: element type of the per-(query, slot) dq partials
 __global__ void k_final_dq(Dims dm, const float* __restrict__ dQacc, const PT* __restrict__ dq_part,
-                           const int32_t* __restrict__ sel, int use_ret, T* __restrict__ dQ) {
+                           const int32_t* __restrict__ sel, const int32_t* __restrict__ bsel, int use_ret, T* __restrict__ dQ) {
   const int pq = blockIdx.y;
   const int t = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), lane = threadIdx.x & 31;
   if (t >= dm.N) return;
@@ -595,11 +602,18 @@ __global__ void k_final_dq(Dims dm, const float* __restrict__ dQacc, const PT* _
 #pragma unroll
   for (int k = 0; k < D / 32; ++k) acc[k] = dQacc[row * D + lane + 32 * k];
   if (use_ret && query_plane_b(dm, t) >= 0) {
+    const int kk = bsel != nullptr ? dm.k2 : 1;            // partial rows per slot: one, or one per chosen block
     for (int s = 0; s < dm.m; ++s) {
       const int c = sel[row * dm.m + s];
       if (c < 0 || c >= dm.Ck) continue;                   // "none", or an entry outside [0, Ck), which counts as none
+      for (int e = 0; e < kk; ++e) {
+        if (bsel != nullptr) {
+          const int bb = bsel[(row * dm.m + s) * kk + e];
+          if (bb < 0 || bb > query_plane_b(dm, t)) continue;
+        }
 #pragma unroll
-      for (int k = 0; k < D / 32; ++k) acc[k] += to_f(dq_part[(row * dm.m + s) * D + lane + 32 * k]);
+        for (int k = 0; k < D / 32; ++k) acc[k] += to_f(dq_part[((row * dm.m + s) * kk + e) * D + lane + 32 * k]);
+      }
     }
   }
 #pragma unroll
@@ -653,6 +667,7 @@ struct BwdWs {
   int32_t *status, *off_q, *perm_q, *sort_scratch, *ret_scratch;
   __nv_bfloat16* qsplit;
   float *delta, *dQacc, *dq_part, *dK_orig, *dV_orig, *dK_perm, *dV_perm, *dkappa, *dnu, *dS;
+  float *dkappa_b, *dnu_b, *dS_b;           // gradients of the per-block summaries (two-level retrieval), fp32
 };
 
 static BwdWs bwd_ws(const Dims& d, Arena& ar) {
@@ -665,7 +680,7 @@ static BwdWs bwd_ws(const Dims& d, Arena& ar) {
   w.ret_scratch = ar.take<int32_t>(pq * ret_index_elems(d));
   w.delta = ar.take<float>(pq * d.N);
   w.dQacc = ar.take<float>(pq * d.N * d.D);
-  w.dq_part = ar.take<float>(pq * d.N * d.m * d.D);
+  w.dq_part = ar.take<float>(pq * d.N * d.m * (d.k2 > 0 ? d.k2 : 1) * d.D);
   w.dK_orig = ar.take<float>(pq * d.N * d.D);
   w.dV_orig = ar.take<float>(pq * d.N * d.D);
   w.dK_perm = ar.take<float>(pq * d.N * d.D);
@@ -674,6 +689,12 @@ static BwdWs bwd_ws(const Dims& d, Arena& ar) {
   w.dnu = ar.take<float>(ent * d.D);
   w.dS = ar.take<float>(ent);
   w.qsplit = ar.take<__nv_bfloat16>(2 * pq * d.Cq * d.D);
+  w.dkappa_b = w.dnu_b = w.dS_b = nullptr;
+  if (d.k2 > 0) {
+    w.dkappa_b = ar.take<float>(ent * d.D);
+    w.dnu_b = ar.take<float>(ent * d.D);
+    w.dS_b = ar.take<float>(ent);
+  }
   return w;
 }
 
@@ -682,10 +703,11 @@ size_t attn_bwd_ws_bytes(const Dims& d, int) { Arena ar(nullptr); bwd_ws(d, ar);
 template <class T, int D>
 static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T* V, const T* O, const float* LSE,
                       const T* dO, const int32_t* assign_q, const float* qbar, const int32_t* off_k,
-                      const int32_t* perm_k, const void* summaries, const int32_t* sel, T* dQ, T* dK, T* dV,
+                      const int32_t* perm_k, const void* summaries, const int32_t* sel, const int32_t* bsel, T* dQ, T* dK, T* dV,
                       void* ws, cudaStream_t st) {
   Arena ar(ws);
   BwdWs w = bwd_ws(d, ar);
+  if (d.k2 == 0) bsel = nullptr;
   const int pq = d.B * d.Hq, pk = d.B * d.Hkv;
   SummLayout L = summ_layout(d, dtype);
   const char* base = (const char*)summaries;
@@ -725,7 +747,7 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
     if (rc != MUSE_OK) return rc;
     if (d.m > 0) {
       RetIndex ri;
-      rc = build_ret_index(d, sel, nullptr, w.ret_scratch, &ri, st);
+      rc = build_ret_index(d, sel, bsel, w.ret_scratch, &ri, st);
       if (rc != MUSE_OK) return rc;
       if (kTensor) {
         rc = ret_bwd_tc(d, Q, dO, Kp, Vp, LSE, w.delta, off_k, ri.goff, ri.pairs, w.dq_part, w.dK_perm, w.dV_perm, w.status, st);
@@ -761,20 +783,38 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
       MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd<T, D, GB>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
       prof_mark("k_summ_bwd", st);
       k_summ_bwd<T, D, GB><<<dim3(d.Ck, pq), kFlashThreads, ssm, st>>>(d, Kp, Vp, off_k, w.off_q, qbar, mu, (const GB*)w.dkappa,
-                                                                     (const GB*)w.dnu, w.dS, w.dK_perm, w.dV_perm);
+                                                                     (const GB*)w.dnu, w.dS, w.dK_perm, w.dV_perm, 0);
     } else {
       MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd<T, D, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
       prof_mark("k_summ_bwd", st);
       k_summ_bwd<T, D, float><<<dim3(d.Ck, pq), kFlashThreads, ssm, st>>>(d, Kp, Vp, off_k, w.off_q, qbar, mu, w.dkappa, w.dnu, w.dS,
-                                                                        w.dK_perm, w.dV_perm);
+                                                                        w.dK_perm, w.dV_perm, 0);
     }
+    MUSE_LAUNCH_OK();
+  }
+  if (d.k2 > 0 && d.m > 0 && d.SB > 0) {
+    // two-level retrieval: the stand-in keys of the non-retrieved blocks of the selected clusters.  Their gradient goes to dQ
+    // directly and to the per-block summaries, from where the key-side pass (per-block mode) carries it to K and V.
+    const size_t ent = (size_t)pq * d.SB * d.Cq * d.Ck;
+    prof_mark("memset", st);
+    MUSE_CUDA_OK(cudaMemsetAsync(w.dkappa_b, 0, ent * d.D * sizeof(float), st));
+    MUSE_CUDA_OK(cudaMemsetAsync(w.dnu_b, 0, ent * d.D * sizeof(float), st));
+    MUSE_CUDA_OK(cudaMemsetAsync(w.dS_b, 0, ent * sizeof(float), st));
+    const SummPtrs spb = summ_ptrs_blk(L, base);
+    int rc = near_bwd(d, dtype, Q, dO, qbar, LSE, w.delta, w.off_q, w.perm_q, sel, bsel, spb, w.dQacc, w.dkappa_b, w.dnu_b, w.dS_b, st);
+    if (rc != MUSE_OK) return rc;
+    const size_t ssm = (size_t)(5 * kTile * (D + 4) + kTile * kLDP) * sizeof(float);
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd<T, D, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
+    prof_mark("k_summ_bwd", st);
+    k_summ_bwd<T, D, float><<<dim3(d.Ck, pq), kFlashThreads, ssm, st>>>(d, Kp, Vp, off_k, w.off_q, qbar, spb.mu, w.dkappa_b, w.dnu_b, w.dS_b,
+                                                                      w.dK_perm, w.dV_perm, 1);
     MUSE_LAUNCH_OK();
   }
   prof_mark("k_final_dq", st);
   if (kTensor)
-    k_final_dq<T, D, __nv_bfloat16><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.dQacc, (const __nv_bfloat16*)w.dq_part, sel, use_ret, dQ);
+    k_final_dq<T, D, __nv_bfloat16><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.dQacc, (const __nv_bfloat16*)w.dq_part, sel, bsel, use_ret, dQ);
   else
-    k_final_dq<T, D, float><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.dQacc, w.dq_part, sel, use_ret, dQ);
+    k_final_dq<T, D, float><<<dim3(cdiv(d.N, 8), pq), 256, 0, st>>>(d, w.dQacc, w.dq_part, sel, bsel, use_ret, dQ);
   MUSE_LAUNCH_OK();
   prof_mark("k_final_dkv", st);
   k_final_dkv<T, D><<<dim3(cdiv(d.N * (D / 4), 256), pk), 256, 0, st>>>(d, perm_k, w.dK_orig, w.dV_orig, w.dK_perm, w.dV_perm,
@@ -785,10 +825,11 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
 
 int attn_bwd(const Dims& d, int dtype, const void* Q, const void* K, const void* V, const void* O, const float* LSE,
              const void* dO, const int32_t* assign_q, const float* qbar, const int32_t* off_k, const int32_t* perm_k,
-             const void* summaries, const int32_t* sel, void* dQ, void* dK, void* dV, void* ws, cudaStream_t st) {
+             const void* summaries, const int32_t* sel, const int32_t* bsel, void* dQ, void* dK, void* dV, void* ws,
+             cudaStream_t st) {
   typedef __nv_bfloat16 bf;
 #define MUSE_BWD(TT, DD) attn_bwd_t<TT, DD>(d, dtype, (const TT*)Q, (const TT*)K, (const TT*)V, (const TT*)O, LSE, (const TT*)dO, \
-                                            assign_q, qbar, off_k, perm_k, summaries, sel, (TT*)dQ, (TT*)dK, (TT*)dV, ws, st)
+                                            assign_q, qbar, off_k, perm_k, summaries, sel, bsel, (TT*)dQ, (TT*)dK, (TT*)dV, ws, st)
   if (dtype == MUSE_F32) return d.D == 64 ? MUSE_BWD(float, 64) : MUSE_BWD(float, 128);
   return d.D == 64 ? MUSE_BWD(bf, 64) : MUSE_BWD(bf, 128);
 #undef MUSE_BWD

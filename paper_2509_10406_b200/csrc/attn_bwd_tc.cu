@@ -775,7 +775,7 @@ int ret_bwd_tc(const Dims& d, const void* Q, const void* dO, const void* Kp, con
                const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, void* dq_part,
                float* dK_perm, float* dV_perm, int* status, cudaStream_t st) {
   const int pq = d.B * d.Hq;
-  if (!path_forced(kForceRetBwdSplit))
+  if (!path_forced(kForceRetBwdSplit) || d.k2 > 0)
     return ret_bwd_pairs_tc(d, Q, dO, Kp, Vp, LSE, delta, off_k, goff, pairs, dq_part, dK_perm, dV_perm, status, st);
   prof_mark("k_ret_bwd_dkdv_tc", st);
   MUSE_TC_LAUNCH(k_ret_bwd_dkdv_tc, KeysSmem, kKeysThreads, dim3(d.Ck, d.SB * kRetSplit, pq), d, (const bf16*)Q, (const bf16*)dO, (const bf16*)Kp,

@@ -233,7 +233,7 @@ size_t attn_fwd_ws_bytes(const Dims& d, int dtype);
 
 int attn_bwd(const Dims& d, int dtype, const void* Q, const void* K, const void* V, const void* O,
              const float* LSE, const void* dO, const int32_t* assign_q, const float* qbar,
-             const int32_t* off_k, const int32_t* perm_k, const void* summaries, const int32_t* sel,
+             const int32_t* off_k, const int32_t* perm_k, const void* summaries, const int32_t* sel, const int32_t* bsel,
              void* dQ, void* dK, void* dV, void* ws, cudaStream_t st);
 size_t attn_bwd_ws_bytes(const Dims& d, int dtype);
 

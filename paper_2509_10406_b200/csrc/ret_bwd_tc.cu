@@ -68,15 +68,19 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   __shared__ int32_t ok_s[kOkCache];
   __shared__ int32_t tok_s[2][kPairs];                      // tokens of the tile each half is gathering
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int j = blockIdx.x, sub = blockIdx.y, pq = blockIdx.z;
+  // With spatial block selection (k2 > 0) the CTA owns one BUCKET (cluster j, block bb): its pairs are the (query, slot,
+  // chosen block) triples that chose the block, and every one of them sees the whole bucket (as in the forward kernel).
+  const bool bucket = dm.k2 > 0;
+  const int j = bucket ? blockIdx.x / dm.SB : blockIdx.x, bb = bucket ? blockIdx.x % dm.SB : 0, sub = blockIdx.y, pq = blockIdx.z;
+  const int mk = dm.m * (bucket ? dm.k2 : 1);               // partial dQ rows per query
   const int b_ = pq / dm.Hq, h = pq % dm.Hq, pk = b_ * dm.Hkv + dm.hm.g[h];
   const int ngroups = dm.SB * dm.Ck;
-  const int32_t* go = goff + (size_t)pq * (ngroups + 1) + (size_t)j * dm.SB;   // the cluster's pairs: plane pl is [go[pl], go[pl + 1])
-  const int g0 = go[0], g1 = go[dm.SB];
+  const int32_t* go = goff + (size_t)pq * (ngroups + 1) + (size_t)j * dm.SB + bb;   // the group's pairs: plane pl is [go[pl], go[pl + 1])
+  const int g0 = go[0], g1 = go[bucket ? 1 : dm.SB];
   const int ntiles = (g1 - g0 + kPairs - 1) / kPairs;
   const int nsub = min(kSplit, max(1, ntiles / kTilesPerCta));            // tiles are dealt round-robin to nsub CTAs
   const int32_t* okg = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;   // okg[b]: first key of bucket (j, b)
-  const int k0 = okg[0], kall = okg[dm.SB] - k0;                          // keys that some plane sees
+  const int k0 = okg[bb], kall = (bucket ? okg[bb + 1] : okg[dm.SB]) - k0;   // keys that some pair of the group sees
   if (ntiles == 0 || sub >= nsub) return;
   if (tc::smem_u32(sm) & 1023u) {                           // the tiles fill the whole dynamic allocation: no room to realign
     if (tid == 0) report_status(status, MUSE_STATUS_BWD_TIMEOUT);
@@ -100,8 +104,8 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   const bf16* dOb = dO + (size_t)pq * dm.N * D;
   const bf16* Kb = Kp + ((size_t)pk * dm.N + k0) * D;
   const bf16* Vb = Vp + ((size_t)pk * dm.N + k0) * D;
-  const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
-  const size_t pbase = (size_t)pq * dm.N * dm.m;
+  const int32_t* pr = pairs + (size_t)pq * dm.N * mk;
+  const size_t pbase = (size_t)pq * dm.N * mk;
   // role of this warp: half v, and row / issuing / gather warp
   const bool roww = warp < 2 * kRowWarps, issw = warp >= kIssuerWarp0 && warp < kIssuerWarp0 + 2, gatw = warp >= kGatherWarp0;
   const int v = roww ? warp / kRowWarps : issw ? warp - kIssuerWarp0 : (warp - kGatherWarp0) / (kGather / 32);
@@ -112,6 +116,7 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
   auto wait = [&](uint64_t* bar, uint32_t parity) { if (ok_ && !tc::mbar_wait(bar, parity)) ok_ = false; };
   // keys of sweep `kc` that the query of pair `pid` sees (its block's prefix of the cluster)
   auto visible = [&](int pid, int kc) {
+    if (bucket) return min(kKeys, max(0, kall - kc));
     const int tok = pid / dm.m;
     return min(kKeys, max(0, ok[dm.causal ? tok / dm.Bs : 1] - k0 - kc));
   };
@@ -131,7 +136,7 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
     const int nkc = max(0, min(kKeys, kall - kc));
     // later sweeps pass over the tiles of planes that see none of the sweep's keys (a prefix of the cluster's tiles)
     int tile_lo = 0;
-    if (!first) {
+    if (!first && !bucket) {
       int pl = 0;
       while (pl + 1 < dm.SB && ok[pl + 1] - k0 <= kc) ++pl;
       tile_lo = (go[pl] - g0) / kPairs;
@@ -164,12 +169,12 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
       auto ld_pid = [&](int t) {
         const int t0 = g0 + t * kPairs;
         const int id = (t < ntiles && t0 + row < g1) ? __ldg(pr + t0 + row) : -1;
-        return id >= 0 && !MUSE_IN_RANGE(id, (long long)dm.N * dm.m) ? -1 : id;
+        return id >= 0 && !MUSE_IN_RANGE(id, (long long)dm.N * mk) ? -1 : id;
       };
       int pid = ld_pid(tile0), pid_n = ld_pid(tile0 + tstep);
       float L2 = 0.f, dl = 0.f, L2_n = 0.f, dl_n = 0.f;
       auto ld_scalars = [&](int p, float& l2, float& d_) {
-        const size_t tt = (size_t)pq * dm.N + max(p, 0) / dm.m;
+        const size_t tt = (size_t)pq * dm.N + max(p, 0) / mk;
         l2 = p >= 0 ? LSE[tt] * kLog2e : 0.f;
         d_ = p >= 0 ? delta[tt] : 0.f;
       };
@@ -345,7 +350,7 @@ k_ret_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const bf16* __restrict__
         RBCLK(0)
         if (np > 0) wait(&B.q_empty, (np - 1) & 1);          // the previous tile's products have read the buffers
         RBCLK(1)
-        tok_s[v][g] = pa_ >= 0 ? pa_ / dm.m : -1;
+        tok_s[v][g] = pa_ >= 0 ? pa_ / mk : -1;
         tc::named_bar_sync(1 + v, kGather);
 #pragma unroll 4
         for (int r = g / (D / 8); r < kPairs; r += RPP) {
@@ -392,7 +397,7 @@ int ret_bwd_pairs_tc(const Dims& d, const void* Q, const void* dO, const void* K
                      const float* delta, const int32_t* off_k, const int32_t* goff, const int32_t* pairs, void* dq_part,
                      float* dK_perm, float* dV_perm, int* status, cudaStream_t st) {
   prof_mark("k_ret_bwd_pairs_tc", st);
-  const dim3 grid(d.Ck, rb::kSplit, d.B * d.Hq);
+  const dim3 grid(d.k2 > 0 ? d.Ck * d.SB : d.Ck, rb::kSplit, d.B * d.Hq);      // one CTA (or a few) per key cluster, or per bucket
   if (d.D == 128) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_ret_bwd_pairs_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, rb::Lay<128>::kSmem));
     k_ret_bwd_pairs_tc<128><<<grid, rb::kThreads, rb::Lay<128>::kSmem, st>>>(

@@ -74,8 +74,12 @@ def test_null_and_small_workspace_are_rejected(mb):
     need = mb.muse_workspace_bytes(p)
     assert need[5] == need[3] + need[4] + need[1]
     a16 = [fake] * 9
-    assert L.muse_attn_bwd(ctypes.byref(p), fake, fake, fake, fake, fake, fake, fake, fake, fake, fake, z, fake,
+    assert L.muse_attn_bwd(ctypes.byref(p), fake, fake, fake, fake, fake, fake, fake, fake, fake, fake, z, fake, z,
                            fake, fake, fake, fake, need[3], z) == -3
+    # two-level retrieval: the backward pass needs the forward's chosen blocks
+    p2 = mb.make_params(B=1, Hq=1, Hkv=1, N=1024, D=64, Cq=8, Ck=16, m=4, k2=1)
+    assert L.muse_attn_bwd(ctypes.byref(p2), fake, fake, fake, fake, fake, fake, fake, fake, fake, fake, fake, fake, z,
+                           fake, fake, fake, fake, 1 << 40, z) == -1
 
 
 def test_head_map(mb):
