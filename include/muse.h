@@ -91,7 +91,7 @@ typedef struct muse_params {
   int32_t k2;                   /* spatial selection inside the selected clusters (Section "Two-Level Retrieval"):
                                    0 = every earlier block is retrieved; 1..8 = only the k2 best-scoring earlier
                                    blocks, the others enter through their per-block summaries (bf16 mode, causal,
-                                   forward only; ignored when !causal)                                           */
+                                   m * k2 <= 64, S - 1 <= 32; ignored when !causal)                              */
   int32_t dtype;                /* MUSE_BF16 | MUSE_F32: type of Q,K,V,O,dO,dQ,dK,dV               */
   float   softmax_scale;        /* sigma; <= 0 -> 1/sqrt(D)                                        */
   int32_t kmeans_iters;         /* T Lloyd iterations before the final assignment (>= 0)           */

@@ -30,7 +30,7 @@ constexpr int kAtThreads = 320, kAtEpi = 256;
 
 struct AtBars { uint64_t full[4], empty[4], tfull[2], tempty[2], xbar; };
 
-template <int D>
+template <int D, bool DIST>     // DIST: also write the matrix |c|^2 - 2 x.c (the balanced assignment's second step reads it)
 __global__ void __launch_bounds__(kAtThreads, 1)
 k_assign_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CUtensorMap tm_hi, const __grid_constant__ CUtensorMap tm_lo,
             int N, int C, int ns, const float* __restrict__ cnorm, int32_t* __restrict__ assign, float* __restrict__ dist_out,
@@ -117,10 +117,12 @@ k_assign_tc(const __grid_constant__ CUtensorMap tm_x, const __grid_constant__ CU
         const int c0 = t * kAtCols + wg * 64 + 32 * q;
 #pragma unroll
         for (int k = 0; k < 32; ++k) {
-          v[k] = fmaf(-2.f, v[k], cn[c0 + k]);
-          if (v[k] < best) { best = v[k]; bidx = c0 + k; }     // ascending index: ties keep the lower
+          const float dist = fmaf(-2.f, v[k], cn[c0 + k]);
+          if (dist < best) { best = dist; bidx = c0 + k; }     // ascending index: ties keep the lower
         }
-        if (dist_out != nullptr && row0 + row < N) {             // optional output: the whole matrix |c|^2 - 2 x.c
+        if (DIST && row0 + row < N) {                            // optional output: the whole matrix |c|^2 - 2 x.c
+#pragma unroll
+          for (int k = 0; k < 32; ++k) v[k] = fmaf(-2.f, v[k], cn[c0 + k]);
           float* dr = dist_out + ((size_t)prob * N + row0 + row) * C + c0;
           if (c0 + 32 <= C && (C & 3) == 0) {
 #pragma unroll
@@ -169,13 +171,14 @@ int assign_tc(const void* X, int problems, int N, int D, int C, const float* cen
   const size_t smem = (size_t)kAtRows * D * 2 + (size_t)ns * 2 * kAtCols * D * 2 + (size_t)NT * kAtCols * 4 + 1024;
   dim3 grid(cdiv(N, kAtRows), problems);
   prof_mark("k_assign_tc", st);
-  if (D == 128) {
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_assign_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_assign_tc<128><<<grid, kAtThreads, smem, st>>>(tx, thi, tlo, N, C, ns, cnorm, assign, dist_out, status);
-  } else {
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_assign_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k_assign_tc<64><<<grid, kAtThreads, smem, st>>>(tx, thi, tlo, N, C, ns, cnorm, assign, dist_out, status);
+#define MUSE_AT_LAUNCH(DD, DI)                                                                                             \
+  {                                                                                                                        \
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_assign_tc<DD, DI>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));      \
+    k_assign_tc<DD, DI><<<grid, kAtThreads, smem, st>>>(tx, thi, tlo, N, C, ns, cnorm, assign, dist_out, status);        \
   }
+  if (D == 128) { if (dist_out) MUSE_AT_LAUNCH(128, true) else MUSE_AT_LAUNCH(128, false) }
+  else { if (dist_out) MUSE_AT_LAUNCH(64, true) else MUSE_AT_LAUNCH(64, false) }
+#undef MUSE_AT_LAUNCH
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }

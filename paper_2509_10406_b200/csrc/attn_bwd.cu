@@ -602,17 +602,24 @@ __global__ void k_final_dq(Dims dm, const float* __restrict__ dQacc, const PT* _
 #pragma unroll
   for (int k = 0; k < D / 32; ++k) acc[k] = dQacc[row * D + lane + 32 * k];
   if (use_ret && query_plane_b(dm, t) >= 0) {
-    const int kk = bsel != nullptr ? dm.k2 : 1;            // partial rows per slot: one, or one per chosen block
-    for (int s = 0; s < dm.m; ++s) {
-      const int c = sel[row * dm.m + s];
-      if (c < 0 || c >= dm.Ck) continue;                   // "none", or an entry outside [0, Ck), which counts as none
-      for (int e = 0; e < kk; ++e) {
-        if (bsel != nullptr) {
-          const int bb = bsel[(row * dm.m + s) * kk + e];
-          if (bb < 0 || bb > query_plane_b(dm, t)) continue;
-        }
+    if (bsel == nullptr) {                                 // one partial row per slot
+      for (int s = 0; s < dm.m; ++s) {
+        const int c = sel[row * dm.m + s];
+        if (c < 0 || c >= dm.Ck) continue;                 // "none", or an entry outside [0, Ck), which counts as none
 #pragma unroll
-        for (int k = 0; k < D / 32; ++k) acc[k] += to_f(dq_part[((row * dm.m + s) * kk + e) * D + lane + 32 * k]);
+        for (int k = 0; k < D / 32; ++k) acc[k] += to_f(dq_part[(row * dm.m + s) * D + lane + 32 * k]);
+      }
+    } else {                                               // two-level retrieval: one per (slot, chosen block)
+      const int kk = dm.k2, pl = query_plane_b(dm, t);
+      for (int s = 0; s < dm.m; ++s) {
+        const int c = sel[row * dm.m + s];
+        if (c < 0 || c >= dm.Ck) continue;
+        for (int e = 0; e < kk; ++e) {
+          const int bb = bsel[(row * dm.m + s) * kk + e];
+          if (bb < 0 || bb > pl) continue;
+#pragma unroll
+          for (int k = 0; k < D / 32; ++k) acc[k] += to_f(dq_part[((row * dm.m + s) * kk + e) * D + lane + 32 * k]);
+        }
       }
     }
   }
