@@ -10,7 +10,8 @@ namespace muse {
 
 int near_bwd(const Dims& d, int dtype, const void* Q, const void* dO, const float* qbar, const float* LSE, const float* delta,
              const int32_t* off_q, const int32_t* perm_q, const int32_t* sel, const int32_t* bsel, const SummPtrs& sp, float* dQacc,
-             float* dkappa_b, float* dnu_b, float* dS_b, cudaStream_t st);
+             float* dkappa_b, float* dnu_b, float* dS_b, int grad_ji, cudaStream_t st);
+int grad_to_bf16(const float* in, size_t n, void* out, cudaStream_t st);
 
 __device__ __forceinline__ int query_plane_b(const Dims& d, int t) { return d.causal ? t / d.Bs - 1 : 0; }
 
@@ -668,7 +669,7 @@ int far_bwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const void* dO,
 bool summ_bwd_tc_supported(const Dims& d, int dtype);
 int summ_bwd_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* off_q, const float* qbar,
                 const float* mu, const void* dkappa, const void* dnu, const float* dS, float* dK_perm, float* dV_perm,
-                void* qsplit, int* status, cudaStream_t st);
+                void* qsplit, int per_block, int* status, cudaStream_t st);
 
 struct BwdWs {
   int32_t *status, *off_q, *perm_q, *sort_scratch, *ret_scratch;
@@ -783,7 +784,7 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
     }
     const size_t ssm = (size_t)(5 * kTile * (D + 4) + kTile * kLDP) * sizeof(float);
     if (summ_tc) {
-      rc = summ_bwd_tc(d, Kp, Vp, off_k, w.off_q, qbar, mu, w.dkappa, w.dnu, w.dS, w.dK_perm, w.dV_perm, w.qsplit, w.status, st);
+      rc = summ_bwd_tc(d, Kp, Vp, off_k, w.off_q, qbar, mu, w.dkappa, w.dnu, w.dS, w.dK_perm, w.dV_perm, w.qsplit, 0, w.status, st);
       if (rc != MUSE_OK) return rc;
     } else if (far_tc) {
       typedef __nv_bfloat16 GB;
@@ -808,14 +809,26 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
     MUSE_CUDA_OK(cudaMemsetAsync(w.dnu_b, 0, ent * d.D * sizeof(float), st));
     MUSE_CUDA_OK(cudaMemsetAsync(w.dS_b, 0, ent * sizeof(float), st));
     const SummPtrs spb = summ_ptrs_blk(L, base);
-    int rc = near_bwd(d, dtype, Q, dO, qbar, LSE, w.delta, w.off_q, w.perm_q, sel, bsel, spb, w.dQacc, w.dkappa_b, w.dnu_b, w.dS_b, st);
+    const bool tcb = summ_bwd_tc_supported(d, dtype) && !path_forced(kForceSummBwdSimt);
+    int rc = near_bwd(d, dtype, Q, dO, qbar, LSE, w.delta, w.off_q, w.perm_q, sel, bsel, spb, w.dQacc, w.dkappa_b, w.dnu_b, w.dS_b,
+                      tcb ? 1 : 0, st);
     if (rc != MUSE_OK) return rc;
-    const size_t ssm = (size_t)(5 * kTile * (D + 4) + kTile * kLDP) * sizeof(float);
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd<T, D, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
-    prof_mark("k_summ_bwd", st);
-    k_summ_bwd<T, D, float><<<dim3(d.Ck, pq), kFlashThreads, ssm, st>>>(d, Kp, Vp, off_k, w.off_q, qbar, spb.mu, w.dkappa_b, w.dnu_b, w.dS_b,
-                                                                      w.dK_perm, w.dV_perm, 1);
-    MUSE_LAUNCH_OK();
+    if (tcb) {
+      // tensor-core key-side kernel in per-block mode: its gradient tiles are bf16, laid out [plane][j][i]; the buffers of the
+      // accumulated-summary gradients have been consumed by now and take the converted copies
+      rc = grad_to_bf16(w.dkappa_b, ent * d.D, w.dkappa, st);
+      if (rc == MUSE_OK) rc = grad_to_bf16(w.dnu_b, ent * d.D, w.dnu, st);
+      if (rc == MUSE_OK)
+        rc = summ_bwd_tc(d, Kp, Vp, off_k, w.off_q, qbar, spb.mu, w.dkappa, w.dnu, w.dS_b, w.dK_perm, w.dV_perm, w.qsplit, 1, w.status, st);
+      if (rc != MUSE_OK) return rc;
+    } else {
+      const size_t ssm = (size_t)(5 * kTile * (D + 4) + kTile * kLDP) * sizeof(float);
+      MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd<T, D, float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssm));
+      prof_mark("k_summ_bwd", st);
+      k_summ_bwd<T, D, float><<<dim3(d.Ck, pq), kFlashThreads, ssm, st>>>(d, Kp, Vp, off_k, w.off_q, qbar, spb.mu, w.dkappa_b, w.dnu_b, w.dS_b,
+                                                                        w.dK_perm, w.dV_perm, 1);
+      MUSE_LAUNCH_OK();
+    }
   }
   prof_mark("k_final_dq", st);
   if (kTensor)

@@ -40,7 +40,8 @@ __global__ void __launch_bounds__(kNbThreads)
 k_near_bwd(Dims dm, const T* __restrict__ Q, const T* __restrict__ dO, const float* __restrict__ qbar, const float* __restrict__ LSE,
            const float* __restrict__ delta, const int32_t* __restrict__ off_q, const int32_t* __restrict__ perm_q,
            const int32_t* __restrict__ sel, const int32_t* __restrict__ bsel, SummPtrs sp, float* __restrict__ dQacc,
-           float* __restrict__ dkappa_b, float* __restrict__ dnu_b, float* __restrict__ dS_b) {
+           float* __restrict__ dkappa_b, float* __restrict__ dnu_b, float* __restrict__ dS_b, int grad_ji) {
+  // grad_ji: the gradient entries are laid out [plane][j][i] (what the tensor-core key-side kernel reads) instead of [plane][i][j]
   constexpr int EPL = D / 32, ROWS = nb_rows<T>();
   extern __shared__ __align__(16) unsigned char nb_smem[];
   const int m = dm.m, k2 = dm.k2, SB = dm.SB, Ck = dm.Ck;
@@ -199,7 +200,7 @@ k_near_bwd(Dims dm, const T* __restrict__ Q, const T* __restrict__ dO, const flo
         if (touched_s) {                                               // (block-uniform) flush into the gradient entries (b', i, j), which this CTA owns
           for (int e = tid; e < b * D; e += kNbThreads) {
             const int bp = e / D, d0 = e % D;
-            const size_t ent = ebase + (size_t)bp * estep + j;
+            const size_t ent = grad_ji ? (((size_t)pq * SB + bp) * Ck + j) * dm.Cq + i : ebase + (size_t)bp * estep + j;
             const float a = gka[e], c = gnu[e];
             if (a != 0.f) dkappa_b[ent * D + d0] += a;
             if (c != 0.f) dnu_b[ent * D + d0] += c;
@@ -207,7 +208,7 @@ k_near_bwd(Dims dm, const T* __restrict__ Q, const T* __restrict__ dO, const flo
           }
           if (tid < b) {
             const float a = gmu[tid];
-            if (a != 0.f) dS_b[ebase + (size_t)tid * estep + j] += a;
+            if (a != 0.f) dS_b[grad_ji ? (((size_t)pq * SB + tid) * Ck + j) * dm.Cq + i : ebase + (size_t)tid * estep + j] += a;
             gmu[tid] = 0.f;
           }
         }
@@ -230,6 +231,21 @@ k_near_bwd(Dims dm, const T* __restrict__ Q, const T* __restrict__ dO, const flo
   }
 }
 
+// fp32 gradient rows -> bf16 (the operand type of the tensor-core key-side kernel), same layout
+__global__ void k_grad_to_bf16(const float* __restrict__ in, long long n4, __nv_bfloat16* __restrict__ out) {
+  const long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= n4) return;
+  st4(out + 4 * e, ld4(in + 4 * e));
+}
+
+int grad_to_bf16(const float* in, size_t n, void* out, cudaStream_t st) {
+  const long long n4 = (long long)(n / 4);
+  prof_mark("k_grad_to_bf16", st);
+  k_grad_to_bf16<<<(unsigned)((n4 + 255) / 256), 256, 0, st>>>(in, n4, (__nv_bfloat16*)out);
+  MUSE_LAUNCH_OK();
+  return MUSE_OK;
+}
+
 size_t near_bwd_smem_bytes(const Dims& d, int elem_bytes) {
   const size_t stage = (size_t)d.SB * (elem_bytes == 2 ? 3 : 2) * d.D * elem_bytes + (size_t)kNbMaxBlocks * sizeof(float);
   return 2 * stage + (size_t)(2 * d.SB * d.D + kNbMaxBlocks) * sizeof(float) + (size_t)kNbChunk * (d.m + 1) * sizeof(int) +
@@ -239,26 +255,26 @@ size_t near_bwd_smem_bytes(const Dims& d, int elem_bytes) {
 template <class T, int D>
 static int near_bwd_t(const Dims& d, const T* Q, const T* dO, const float* qbar, const float* LSE, const float* delta,
                       const int32_t* off_q, const int32_t* perm_q, const int32_t* sel, const int32_t* bsel, const SummPtrs& sp,
-                      float* dQacc, float* dkappa_b, float* dnu_b, float* dS_b, cudaStream_t st) {
+                      float* dQacc, float* dkappa_b, float* dnu_b, float* dS_b, int grad_ji, cudaStream_t st) {
   const size_t smem = near_bwd_smem_bytes(d, (int)sizeof(T));
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_near_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prof_mark("k_near_bwd", st);
   k_near_bwd<T, D><<<dim3(d.Cq, d.B * d.Hq), kNbThreads, smem, st>>>(d, Q, dO, qbar, LSE, delta, off_q, perm_q, sel, bsel, sp, dQacc,
-                                                                   dkappa_b, dnu_b, dS_b);
+                                                                   dkappa_b, dnu_b, dS_b, grad_ji);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }
 
 int near_bwd(const Dims& d, int dtype, const void* Q, const void* dO, const float* qbar, const float* LSE, const float* delta,
              const int32_t* off_q, const int32_t* perm_q, const int32_t* sel, const int32_t* bsel, const SummPtrs& sp, float* dQacc,
-             float* dkappa_b, float* dnu_b, float* dS_b, cudaStream_t st) {
+             float* dkappa_b, float* dnu_b, float* dS_b, int grad_ji, cudaStream_t st) {
   typedef __nv_bfloat16 bf;
   if (dtype == MUSE_F32) {
-    if (d.D == 64) return near_bwd_t<float, 64>(d, (const float*)Q, (const float*)dO, qbar, LSE, delta, off_q, perm_q, sel, bsel, sp, dQacc, dkappa_b, dnu_b, dS_b, st);
-    return near_bwd_t<float, 128>(d, (const float*)Q, (const float*)dO, qbar, LSE, delta, off_q, perm_q, sel, bsel, sp, dQacc, dkappa_b, dnu_b, dS_b, st);
+    if (d.D == 64) return near_bwd_t<float, 64>(d, (const float*)Q, (const float*)dO, qbar, LSE, delta, off_q, perm_q, sel, bsel, sp, dQacc, dkappa_b, dnu_b, dS_b, grad_ji, st);
+    return near_bwd_t<float, 128>(d, (const float*)Q, (const float*)dO, qbar, LSE, delta, off_q, perm_q, sel, bsel, sp, dQacc, dkappa_b, dnu_b, dS_b, grad_ji, st);
   }
-  if (d.D == 64) return near_bwd_t<bf, 64>(d, (const bf*)Q, (const bf*)dO, qbar, LSE, delta, off_q, perm_q, sel, bsel, sp, dQacc, dkappa_b, dnu_b, dS_b, st);
-  return near_bwd_t<bf, 128>(d, (const bf*)Q, (const bf*)dO, qbar, LSE, delta, off_q, perm_q, sel, bsel, sp, dQacc, dkappa_b, dnu_b, dS_b, st);
+  if (d.D == 64) return near_bwd_t<bf, 64>(d, (const bf*)Q, (const bf*)dO, qbar, LSE, delta, off_q, perm_q, sel, bsel, sp, dQacc, dkappa_b, dnu_b, dS_b, grad_ji, st);
+  return near_bwd_t<bf, 128>(d, (const bf*)Q, (const bf*)dO, qbar, LSE, delta, off_q, perm_q, sel, bsel, sp, dQacc, dkappa_b, dnu_b, dS_b, grad_ji, st);
 }
 
 }  // namespace muse

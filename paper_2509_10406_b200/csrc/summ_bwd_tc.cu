@@ -44,7 +44,10 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
               const __grid_constant__ CUtensorMap tm_qhi, const __grid_constant__ CUtensorMap tm_qlo,
               const int32_t* __restrict__ off_k, const int32_t* __restrict__ off_q,
               const float* __restrict__ mu, const float* __restrict__ dS, float* __restrict__ dK_perm,
-              float* __restrict__ dV_perm, int* __restrict__ status) {
+              float* __restrict__ dV_perm, int per_block, int* __restrict__ status) {
+  // per_block = 1 (two-level retrieval): mu and the gradients belong to the PER-BLOCK summaries, plane pl holds the summary
+  // of bucket pl alone; a key chunk then meets only the planes whose bucket it overlaps, and the weights of a plane are
+  // masked to that bucket's keys.
   using namespace sb;
   typedef Lay<D> LY;
   constexpr int kTile = LY::kTile, kKeys = LY::kKeys, oQhi = LY::oQhi, oQlo = LY::oQlo, oDka0 = LY::oDka0, oDnu0 = LY::oDnu0,
@@ -94,8 +97,10 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         tc::tma_load_2d(sm + oV + g * NU * 128, &tm_V, 64 * g, row, &bar_kv);
       }
     }
-    int pl0 = 0;                                          // planes [pl0, SB) see this chunk (bucket ends grow with the plane)
+    int pl0 = 0;                                          // planes [pl0, pl_end) see this chunk (bucket ends grow with the plane)
     while (pl0 < dm.SB && ok_[pl0 + 1] <= c0) ++pl0;
+    int pl_end = dm.SB;
+    if (per_block) { pl_end = pl0; while (pl_end < dm.SB && ok_[pl_end] < c0 + NU) ++pl_end; }
     if (!tc::mbar_wait(&bar_kv, ph_kv)) ok = false;
     ph_kv ^= 1;
     bool started = false;                                 // dK^T / dV^T accumulate in TMEM over all (i tile, plane)
@@ -123,13 +128,14 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
           tc::tma_load_2d(sm + oQhi + g * TI * 128, &tm_qhi, 64 * g, r, &bar_q);
           tc::tma_load_2d(sm + oQlo + g * TI * 128, &tm_qlo, 64 * g, r, &bar_q);
         }
-        if (pl0 < dm.SB) issue_grad(pl0, 0);
+        if (pl0 < pl_end) issue_grad(pl0, 0);
       }
       // which planes hold a non-empty segment of query cluster i (others were never written by the far-field pass)
       uint32_t livemask = 0u;
-      for (int pl = pl0; pl < dm.SB; ++pl) {
+      for (int pl = pl0; pl < pl_end; ++pl) {
         const int blk = dm.causal ? pl + 1 : 0;
-        if (in_range && oq[(size_t)blk * dm.Cq + i + 1] > oq[(size_t)blk * dm.Cq + i]) livemask |= 1u << pl;
+        // (per-block gradients are zero-filled before they are accumulated: every plane's rows are valid)
+        if (in_range && (per_block || oq[(size_t)blk * dm.Cq + i + 1] > oq[(size_t)blk * dm.Cq + i])) livemask |= 1u << pl;
       }
       // tilt logits l_iu = sigma qbar_i . k_u, the same for every plane: once per centroid tile
       if (tid == ISSUER) {
@@ -162,15 +168,16 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
       auto ent_of = [&](int pl) { return (((size_t)pq * dm.SB + pl) * dm.Cq + ic) * dm.Ck + j; };        // summaries: [plane][i][j]
       auto gent_of = [&](int pl) { return (((size_t)pq * dm.SB + pl) * dm.Ck + j) * dm.Cq + ic; };      // gradients: [plane][j][i]
       float mu_n = 0.f, dS_n = 0.f;
-      if (pl0 < dm.SB && ((livemask >> pl0) & 1u)) { mu_n = mu[ent_of(pl0)]; dS_n = dS[gent_of(pl0)]; }
-      for (int pl = pl0, k = 0; pl < dm.SB && ok; ++pl, ++k) {
+      if (pl0 < pl_end && ((livemask >> pl0) & 1u)) { mu_n = mu[ent_of(pl0)]; dS_n = dS[gent_of(pl0)]; }
+      for (int pl = pl0, k = 0; pl < pl_end && ok; ++pl, ++k) {
         const int buf = k & 1;
         const int nk = min(NU, ok_[pl + 1] - c0);
+        const int klo = per_block ? max(0, ok_[pl] - c0) : 0;      // first key of the chunk that this plane weighs
         const bool live = (livemask >> pl) & 1u;
         const float mu_i = mu_n * 1.4426950408889634f, dS_i = dS_n;
         const int oDka = buf ? oQlo : oDka0, oDnu = buf ? oDnu1 : oDnu0;
         const uint32_t aDka = tc::smem_u32(sm + oDka), aDnu = tc::smem_u32(sm + oDnu);
-        if (pl + 1 < dm.SB && ((livemask >> (pl + 1)) & 1u)) { mu_n = mu[ent_of(pl + 1)]; dS_n = dS[gent_of(pl + 1)]; }
+        if (pl + 1 < pl_end && ((livemask >> (pl + 1)) & 1u)) { mu_n = mu[ent_of(pl + 1)]; dS_n = dS[gent_of(pl + 1)]; }
         // The far-field pass wrote every row of the gradient tensors (zeros for an empty segment), so the
         // tiles go to the tensor cores as they land.  The D-contractions of this plane do not depend on the
         // previous plane's i-contractions: they are issued first, and only the W / Wc tiles and the other
@@ -189,7 +196,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
                             tc::smem_desc_sw128(aV + (ks / 4) * NU * 128 + (ks % 4) * 32, 16, 1024), idesc, ks > 0);
           tc::mma_commit(&bar1);
           if (k > 0 && !tc::mbar_wait(&bar2, ph2)) ok = false;      // the previous plane's MMAs are done with the other buffer
-          if (pl + 1 < dm.SB && ok) issue_grad(pl + 1, buf ^ 1);
+          if (pl + 1 < pl_end && ok) issue_grad(pl + 1, buf ^ 1);
         }
         ph_g[buf] ^= 1;
         PCLK(1)
@@ -205,8 +212,8 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
 #pragma unroll
           for (int c = 0; c < 32; c += 2) {
             float w0 = 0.f, w1 = 0.f, c0_ = 0.f, c1_ = 0.f;
-            if (live && 32 * wg + c < nk) { w0 = tc::fast_exp2(lg[c] - mu_i); c0_ = w0 * (dS_i + x1[c] + x2[c]); }
-            if (live && 32 * wg + c + 1 < nk) { w1 = tc::fast_exp2(lg[c + 1] - mu_i); c1_ = w1 * (dS_i + x1[c + 1] + x2[c + 1]); }
+            if (live && 32 * wg + c < nk && 32 * wg + c >= klo) { w0 = tc::fast_exp2(lg[c] - mu_i); c0_ = w0 * (dS_i + x1[c] + x2[c]); }
+            if (live && 32 * wg + c + 1 < nk && 32 * wg + c + 1 >= klo) { w1 = tc::fast_exp2(lg[c + 1] - mu_i); c1_ = w1 * (dS_i + x1[c + 1] + x2[c + 1]); }
             __nv_bfloat162 a = __floats2bfloat162_rn(w0, w1), b = __floats2bfloat162_rn(c0_, c1_);
             ww[c >> 1] = *reinterpret_cast<uint32_t*>(&a); wc[c >> 1] = *reinterpret_cast<uint32_t*>(&b);
           }
@@ -249,7 +256,7 @@ k_summ_bwd_tc(Dims dm, const __grid_constant__ CUtensorMap tm_dka, const __grid_
         pc[6] += 1;
 #endif
       }
-      if (pl0 < dm.SB) {                                  // last plane's MMAs
+      if (pl0 < pl_end) {                                 // last plane's MMAs
         if (!tc::mbar_wait(&bar2, ph2)) ok = false;
         ph2 ^= 1;
         tc::fence_after_sync();
@@ -292,7 +299,7 @@ int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t
 
 int summ_bwd_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* off_q, const float* qbar,
                 const float* mu, const void* dkappa, const void* dnu, const float* dS, float* dK_perm, float* dV_perm,
-                void* qsplit, int* status, cudaStream_t st) {
+                void* qsplit, int per_block, int* status, cudaStream_t st) {
   // qsplit: 2 * B*Hq*Cq*D bf16 of scratch for the split centroids
   bf16* qhi = (bf16*)qsplit;
   bf16* qlo = qhi + (size_t)d.B * d.Hq * d.Cq * d.D;
@@ -313,11 +320,11 @@ int summ_bwd_tc(const Dims& d, const void* Kp, const void* Vp, const int32_t* of
   if (d.D == 128) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb::Lay<128>::total));
     k_summ_bwd_tc<128><<<dim3(d.Ck, d.B * d.Hq), sb::THREADS, sb::Lay<128>::total, st>>>(d, tdka, tdnu, tK, tV, tqh, tql, off_k, off_q, mu, dS,
-                                                                                    dK_perm, dV_perm, status);
+                                                                                    dK_perm, dV_perm, per_block, status);
   } else {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_summ_bwd_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, sb::Lay<64>::total));
     k_summ_bwd_tc<64><<<dim3(d.Ck, d.B * d.Hq), sb::THREADS, sb::Lay<64>::total, st>>>(d, tdka, tdnu, tK, tV, tqh, tql, off_k, off_q, mu, dS,
-                                                                                  dK_perm, dV_perm, status);
+                                                                                  dK_perm, dV_perm, per_block, status);
   }
   MUSE_LAUNCH_OK();
   return MUSE_OK;

@@ -115,8 +115,9 @@ def test_retrieving_every_block_equals_single_level():
     assert np.abs(outs[1][1] - outs[0][1]).max() <= 1e-3 * max(1.0, np.abs(outs[0][1]).max())
 
 
-@pytest.mark.parametrize("name,k2,agg", [("d128", 1, True), ("d128", 2, True), ("tc_d64", 1, True), ("tc", 1, False), ("tc_gqa4", 2, True)])
-def test_two_level_backward_matches_oracle(name, k2, agg):
+@pytest.mark.parametrize("name,k2,agg,force", [("d128", 1, True, 0), ("d128", 2, True, 0), ("tc_d64", 1, True, 0), ("tc", 1, False, 0),
+                                               ("tc_gqa4", 2, True, 0), ("tc", 1, True, 4), ("tc_d64", 2, False, 4)])
+def test_two_level_backward_matches_oracle(name, k2, agg, force):
     """Backward with k2 > 0: the chosen clusters and blocks of the forward pass are constants; dQ, dK, dV against the oracle's
     backward evaluated on the same selections (bf16 mode, 2e-2 relative max-abs)."""
     from paper_2509_10406_b200 import binding as mb
@@ -127,23 +128,28 @@ def test_two_level_backward_matches_oracle(name, k2, agg):
     buf = mb.MuseBuffers(p, backward=True)
     Q, K, V, dO = c.dev()
     aq, qb = to_dev(c.a_q, "i"), to_dev(qbar32, "f32")
-    with kernels_launched() as rec:
-        mb.muse_summarize(p, K, V, to_dev(c.a_k, "i"), qb, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
-        mb.muse_attn_fwd(p, Q, K, V, aq, qb, buf.off_k, buf.perm_k, buf.summaries, None, buf.O, buf.LSE, buf.sel, buf.ws, bsel_out=buf.bsel)
-        torch.cuda.synchronize()
-        assert mb.muse_status(buf.ws) == 0
-        mb.muse_attn_bwd(p, Q, K, V, buf.O, buf.LSE, dO, aq, qb, buf.off_k, buf.perm_k, buf.summaries, buf.sel, buf.dQ, buf.dK, buf.dV,
-                         buf.ws, bsel=buf.bsel)
-        torch.cuda.synchronize()
+    mb.muse_test_force_paths(force)        # 4: the key-side passes (accumulated and per-block) on the FFMA kernel
+    try:
+        with kernels_launched() as rec:
+            mb.muse_summarize(p, K, V, to_dev(c.a_k, "i"), qb, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
+            mb.muse_attn_fwd(p, Q, K, V, aq, qb, buf.off_k, buf.perm_k, buf.summaries, None, buf.O, buf.LSE, buf.sel, buf.ws, bsel_out=buf.bsel)
+            torch.cuda.synchronize()
+            assert mb.muse_status(buf.ws) == 0
+            mb.muse_attn_bwd(p, Q, K, V, buf.O, buf.LSE, dO, aq, qb, buf.off_k, buf.perm_k, buf.summaries, buf.sel, buf.dQ, buf.dK, buf.dV,
+                             buf.ws, bsel=buf.bsel)
+            torch.cuda.synchronize()
+    finally:
+        mb.muse_test_force_paths(0)
     assert mb.muse_status(buf.ws) == 0
-    assert {"k_near_bwd", "k_ret_bwd_pairs_tc", "k_summ_bwd"} <= rec.names, sorted(rec.names)
+    assert {"k_near_bwd", "k_ret_bwd_pairs_tc"} <= rec.names, sorted(rec.names)
+    assert ("k_summ_bwd" in rec.names) == (force == 4) and ("k_grad_to_bf16" in rec.names) == (force == 0), sorted(rec.names)
     sel, bsel = to_np(buf.sel)[..., :w.m], to_np(buf.bsel)
     assert (bsel >= 0).any()
     ref = orc.layer_backward(c.Q.astype(np.float64), c.K.astype(np.float64), c.V.astype(np.float64), c.dO.astype(np.float64),
                              c.a_q, c.a_k, qbar32.astype(np.float64), sigma=c.sigma, S=w.S, Ck=w.Ck, m=w.m, causal=True,
                              sel=sel, sel_mode=0, agg_grad=agg, k2=k2, bsel=bsel)
     errs = dict(dQ=rel_err(to_np(buf.dQ), ref[0]), dK=rel_err(to_np(buf.dK), ref[1]), dV=rel_err(to_np(buf.dV), ref[2]))
-    print(f"[{name} k2={k2} agg={agg}] backward errors {errs}")
+    print(f"[{name} k2={k2} agg={agg} force={force}] backward errors {errs}")
     assert all(v <= tol(w.dtype) for v in errs.values()), errs
     # the near-field term is not negligible in this case: dropping it (the single-level formulas on the same selections)
     # would not pass
