@@ -157,3 +157,26 @@ def test_two_level_backward_matches_oracle(name, k2, agg, force):
                               c.a_q, c.a_k, qbar32.astype(np.float64), sigma=c.sigma, S=w.S, Ck=w.Ck, m=w.m, causal=True,
                               sel=sel, sel_mode=0, agg_grad=agg)
     print("   distance of the single-level gradients:", {k: rel_err(ref0[i], ref[i]) for i, k in enumerate(("dQ", "dK", "dV"))})
+
+
+def test_two_level_backward_rebuilds_both_summary_sets_when_not_given():
+    """summaries = NULL with k2 > 0: the backward pass rebuilds the accumulated AND the per-block summaries in its scratch
+    and returns the same gradients as with the caller's copy (dQ bit for bit; dK, dV end in float atomics)."""
+    from paper_2509_10406_b200 import binding as mb
+    w = TC["tc"]
+    c = Case(w, gain=128.0)
+    qbar32 = c.qbar.astype(np.float32)
+    p = c.params(k2=1)
+    buf = mb.MuseBuffers(p, backward=True)
+    Q, K, V, dO = c.dev()
+    aq, qb = to_dev(c.a_q, "i"), to_dev(qbar32, "f32")
+    mb.muse_summarize(p, K, V, to_dev(c.a_k, "i"), qb, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
+    mb.muse_attn_fwd(p, Q, K, V, aq, qb, buf.off_k, buf.perm_k, buf.summaries, None, buf.O, buf.LSE, buf.sel, buf.ws, bsel_out=buf.bsel)
+    outs = []
+    for summ, ws in ((buf.summaries, buf.ws), (None, torch.empty(buf.sizes[5], dtype=torch.uint8, device="cuda"))):
+        mb.muse_attn_bwd(p, Q, K, V, buf.O, buf.LSE, dO, aq, qb, buf.off_k, buf.perm_k, summ, buf.sel, buf.dQ, buf.dK, buf.dV, ws, bsel=buf.bsel)
+        torch.cuda.synchronize()
+        assert mb.muse_status(ws) == 0
+        outs.append((to_np(buf.dQ), to_np(buf.dK), to_np(buf.dV)))
+    assert np.array_equal(outs[0][0], outs[1][0])
+    assert rel_err(outs[1][1], outs[0][1]) <= 1e-2 and rel_err(outs[1][2], outs[0][2]) <= 1e-2
