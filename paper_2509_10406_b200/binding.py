@@ -29,7 +29,7 @@ EXPORTS = ("muse_workspace_bytes", "muse_summaries_layout", "muse_cluster", "mus
 
 # bits of muse_test_force_paths
 FORCE_SUMM_FWD_SIMT, FORCE_FAR_SIMT, FORCE_SUMM_BWD_SIMT, FORCE_RET_FWD_STREAM = 1, 2, 4, 8
-FORCE_RET_BWD_SPLIT, FORCE_DIPOLE_SIMT = 16, 32
+FORCE_RET_BWD_SPLIT, FORCE_DIPOLE_SIMT, FORCE_BLOCK_SELECT_WARP = 16, 32, 64
 
 
 class MuseParams(ctypes.Structure):

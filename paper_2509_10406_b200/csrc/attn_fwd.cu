@@ -15,6 +15,9 @@ int far_fwd_tc(const Dims& d, const SummPtrs& sp, const void* Q, const int32_t* 
                const int32_t* sel_in, int32_t* sel_out, float* o_far, float* lse_far, int* status, cudaStream_t st);
 int ret_fwd_tc(const Dims& d, const void* Q, const void* Kp, const void* Vp, const int32_t* off_k, const int32_t* goff,
                const int32_t* pairs, void* o_part, float* l_part, int* status, cudaStream_t st);
+bool block_select_q_supported(const Dims& d, int dtype);
+int block_select_q(const Dims& d, const void* Q, const int32_t* off_q, const int32_t* perm_q, const int32_t* sel, const SummPtrs& sp,
+                   const int32_t* bsel_in, int32_t* bsel_out, float* o_near, float* lse_near, int* status, cudaStream_t st);
 int block_select(const Dims& d, int dtype, const void* Q, const int32_t* off_q, const int32_t* perm_q, const int32_t* sel,
                  const SummPtrs& sp, const int32_t* bsel_in, int32_t* bsel_out, float* o_near, float* lse_near, cudaStream_t st);
 
@@ -622,6 +625,9 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
     }
     if (two_level) {
       // second level: the k2 best earlier blocks of every selected cluster, and the near field of the others
+      if (block_select_q_supported(d, dtype) && !path_forced(kForceBlockSelectWarp))
+        rc = block_select_q(d, Q, w.off_q, w.perm_q, sel, summ_ptrs_blk(L, base), bsel_in, bsel, w.o_near, w.lse_near, w.status, st);
+      else
       rc = block_select(d, dtype, Q, w.off_q, w.perm_q, sel, summ_ptrs_blk(L, base), bsel_in, bsel, w.o_near, w.lse_near, st);
       if (rc != MUSE_OK) return rc;
     }

@@ -136,7 +136,7 @@ __device__ __forceinline__ bool dbg_in_range(long long v, long long n, int line)
 // the tensor-core kernel (muse_test_force_paths; never set in production).
 enum ForcePath : unsigned {
   kForceSummFwdSimt = 1u, kForceFarSimt = 2u, kForceSummBwdSimt = 4u, kForceRetFwdStream = 8u,
-  kForceRetBwdSplit = 16u, kForceDipoleSimt = 32u
+  kForceRetBwdSplit = 16u, kForceDipoleSimt = 32u, kForceBlockSelectWarp = 64u
 };
 bool path_forced(unsigned bit);
 

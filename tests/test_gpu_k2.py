@@ -25,10 +25,20 @@ def _run(mb, c, p, buf, Q, K, V, qbar32, sel_in=None, bsel_in=None):
     return to_np(buf.O), to_np(buf.LSE), to_np(buf.sel)[..., :c.w.m], to_np(buf.bsel)
 
 
-@pytest.mark.parametrize("name", list(K2_CASES))
+@pytest.mark.parametrize("name,force", [(n, 0) for n in K2_CASES] + [("tc", 64)])
 @pytest.mark.parametrize("k2", [1, 2])
-def test_two_level_forward_matches_oracle(name, k2):
+def test_two_level_forward_matches_oracle(name, k2, force):
+    """force = 64: the block selection kernel with a warp per query (the one for more than 8 earlier blocks) at a shape where
+    the lane-per-query kernel is the default."""
     from paper_2509_10406_b200 import binding as mb
+    mb.muse_test_force_paths(force)
+    try:
+        _two_level_forward(mb, name, k2, force)
+    finally:
+        mb.muse_test_force_paths(0)
+
+
+def _two_level_forward(mb, name, k2, force):
     w = K2_CASES[name]
     c = Case(w, gain=128.0)
     qbar32 = c.qbar.astype(np.float32)
@@ -38,7 +48,7 @@ def test_two_level_forward_matches_oracle(name, k2):
     with kernels_launched() as rec:
         mb.muse_summarize(p, K, V, to_dev(c.a_k, "i"), to_dev(qbar32, "f32"), buf.off_k, buf.perm_k, buf.summaries, buf.ws)
         O_free, L_free, sel_gpu, bsel_gpu = _run(mb, c, p, buf, Q, K, V, qbar32)
-    assert {"k_block_select", "k_ret_fwd_pairs_tc"} <= rec.names, sorted(rec.names)
+    assert {"k_block_select" if force == 64 else "k_block_select_q", "k_ret_fwd_pairs_tc"} <= rec.names, sorted(rec.names)
     t = tol(w.dtype)
     kw = dict(sigma=c.sigma, S=w.S, Ck=w.Ck, m=w.m, k2=k2)
     sel_orc = np.full((w.B, w.Hq, w.N, w.m), -1, np.int32)
