@@ -40,7 +40,11 @@ backward vs central finite differences with clusters and blocks held fixed, and 
 single-level backward.  Dipole: the Jacobian
 of the far field at zero residual equals the dense-attention Jacobian (a
 cross-covariance written separately in the test), the error falls from first
-to second order in the residual, causality and key-translation invariance.  Streaming k-means: closed-form
+to second order in the residual, causality and key-translation invariance; a covariance tilted at a
+point is the derivative of the tilted value mean at that point (central differences); with retrieval
+(m > 0) the Jacobian at zero residual is still the dense one and the correction is the merge over the
+clusters that were not retrieved; its backward vs central finite differences.  k-means++ seeding: draw
+frequencies against D^2 / sum D^2, distinct indices, one start per separated blob.  Streaming k-means: closed-form
 exponentially weighted means for one cluster and for separated blobs, a hand-computed case that tells
 minibatch assignment from immediate updates, continuation from a saved state; balanced assignment: equals
 the nearest centroid when the cap does not bind, hand-computed overflow cases, size and placement invariants.
@@ -53,7 +57,8 @@ __all__ = [
     "lloyd", "assign_nearest", "assignment_gaps", "strided_init", "feistel_permute",
     "block_summaries", "accumulate", "accumulated_summaries",
     "select_clusters", "forward", "backward", "layer_forward", "layer_backward",
-    "untilted_covariances", "merged_dipole",
+    "untilted_covariances", "tilted_covariances", "mean_query_centroid", "merged_dipole", "dipole_weights",
+    "kmeanspp_init", "kmeanspp_step",
     "stream_order", "streaming_kmeans", "balanced_cap", "balanced_assign",
 ]
 
@@ -140,6 +145,40 @@ def strided_init(N: int, C: int, seed: int, stream: int) -> np.ndarray:
     bijection above: index r -> position pi(r * floor(N/C))."""
     stride = N // C
     return np.array([feistel_permute(r * stride, N, seed, stream) for r in range(C)], np.int32)
+
+
+def _kpp_uniforms(N: int, c: int, seed: int, stream: int) -> np.ndarray:
+    """The N uniforms in (0, 1) of draw number c: integer hash of (seed, stream, c, t) -> 23 bits,
+    centred in their cell, so that every value is exact in single and double precision alike."""
+    key = _splitmix64((seed ^ (stream << 32) ^ (0xA5 << 56) ^ c) & _M64)
+    return np.array([((_splitmix64(key ^ t) >> 41) + 0.5) / 8388608.0 for t in range(N)])
+
+
+def kmeanspp_step(d2, c: int, seed: int, stream: int):
+    """Draw number c (c >= 1) of k-means++ seeding: one index with probability proportional to d2
+    (squared distance to the nearest start point chosen so far).  The draw is an exponential race:
+    every point gets e_t = -log(u_t) from its own uniform and the largest d2_t / e_t wins (lowest
+    index on exact ties), which selects t with probability d2_t / sum(d2) and needs no prefix sum.
+    If every distance is zero the lowest index wins.  Returns (index, race keys)."""
+    d2 = np.asarray(d2, np.float64)
+    e = -np.log(_kpp_uniforms(d2.shape[0], c, seed, stream))
+    keys = d2 / e
+    return int(np.argmax(keys)), keys
+
+
+def kmeanspp_init(X, C: int, seed: int, stream: int) -> np.ndarray:
+    """Seeded k-means++ start indices (plain, one candidate per draw): the first is position 0 of the
+    seeded shuffle, each further one is drawn by kmeanspp_step from the squared distances to the
+    nearest start point so far."""
+    X = np.asarray(X, np.float64)
+    N = X.shape[0]
+    idx = [feistel_permute(0, N, seed, stream)]
+    d2 = ((X - X[idx[0]]) ** 2).sum(1)
+    for c in range(1, C):
+        nxt, _ = kmeanspp_step(d2, c, seed, stream)
+        idx.append(nxt)
+        d2 = np.minimum(d2, ((X - X[nxt]) ** 2).sum(1))
+    return np.asarray(idx, np.int32)
 
 
 # --------------------------------------------------------------------------------------------
@@ -327,6 +366,52 @@ def untilted_covariances(K, V, a_k, S, Ck, causal=True):
     return cov
 
 
+def mean_query_centroid(qbar, a_q):
+    """qbar_star: the mean of the query centroids weighted by the number of queries each holds
+    (the single shared tilt point of "Untilted (Partially Specialized) Covariances")."""
+    qbar = np.asarray(qbar, np.float64)
+    n = np.bincount(np.asarray(a_q, np.int64), minlength=qbar.shape[0]).astype(np.float64)
+    return (n[:, None] * qbar).sum(0) / n.sum()
+
+
+def tilted_covariances(K, V, a_k, S, Ck, tilt, sigma, causal=True):
+    """Shared covariance with one tilt point: as untilted_covariances, but the members of M_jb carry
+    the weights w_u proportional to exp(sigma tilt . k_u), normalised inside the set:
+    Cov_jb = sum_u w_u v_u k_u^T - (sum_u w_u v_u)(sum_u w_u k_u)^T.  tilt = 0 is the untilted case."""
+    K = np.asarray(K, np.float64); V = np.asarray(V, np.float64); tilt = np.asarray(tilt, np.float64)
+    N, D = K.shape; Dv = V.shape[1]
+    if not causal:
+        S = 1
+    Bs = N // S
+    blk = np.arange(N) // Bs
+    cov = np.zeros((S, Ck, Dv, D))
+    for b in range(S):
+        vis = (blk < b) if causal else np.ones(N, bool)
+        for j in range(Ck):
+            mem = np.nonzero(vis & (a_k == j))[0]
+            if mem.size == 0:
+                continue
+            k, v = K[mem], V[mem]
+            l = sigma * (k @ tilt)
+            w = np.exp(l - l.max()); w /= w.sum()
+            cov[b, j] = (w[:, None] * v).T @ k - np.outer(w @ v, w @ k)
+    return cov
+
+
+def dipole_weights(muh):
+    """Centroid attention weights p_ib(j) = softmax_j muh_ijb over the non-empty key clusters
+    (zero elsewhere, and all zero where nothing is visible).  muh [S,Cq,Ck] -> [S,Cq,Ck]."""
+    p = np.zeros_like(muh)
+    S, Cq, _ = muh.shape
+    for b in range(S):
+        for i in range(Cq):
+            fin = np.isfinite(muh[b, i])
+            if fin.any():
+                e = np.where(fin, np.exp(np.where(fin, muh[b, i], 0.0) - muh[b, i][fin].max()), 0.0)
+                p[b, i] = e / e.sum()
+    return p
+
+
 def merged_dipole(muh, cov):
     """Pre-merged dipole matrix per query cluster and block: Cbar_ib = sum_j p_ib(j) Cov_0jb
     with the centroid attention weights p_ib(j) = softmax_j muh_ijb over the non-empty key
@@ -395,12 +480,16 @@ def select_blocks(bl, k2):
 
 
 def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs, m, causal,
-             sel_rows, sel_mode, cbar_ib=None, k2=0, blk_i=None, bsel_rows=None):
+             sel_rows, sel_mode, cbar_ib=None, k2=0, blk_i=None, bsel_rows=None, dip=None):
     """All quantities of Algorithm 1's per-query loop for the queries `rows`, which share the
     query cluster (centroid qbar_i) and the spatial block b.
     k2 > 0 (Section "Two-Level Retrieval", spatial block selection): inside every selected cluster
     only the k2 best-scoring earlier blocks are retrieved exactly; its other earlier blocks enter
-    through their PER-BLOCK summaries `blk_i` = (mu, kappa, nu)[b', j] of this query cluster."""
+    through their PER-BLOCK summaries `blk_i` = (mu, kappa, nu)[b', j] of this query cluster.
+    `dip` = (p_ib [Ck], cov_b [Ck,Dv,D]): dipole correction next to retrieval (Appendix "Compatibility
+    with Retrieval"): the retrieved clusters are attended exactly, so their share leaves the merged
+    matrix -- the correction of a query is the merge over the clusters it did NOT retrieve, with the
+    centroid weights renormalised over those: (sum_{j far} p(j) Cov_jb) qres / sum_{j far} p(j)."""
     N = K.shape[0]
     Ck = muh_ib.shape[0]
     qp = sigma * Q[rows]                                   # full (scaled) query
@@ -428,6 +517,15 @@ def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs
     if cbar_ib is not None:
         # dipole: the linear value term, merged over clusters; the mass (lse_far) is unchanged
         o_far = o_far + np.where(np.isfinite(lse_far)[:, None], qres @ cbar_ib.T, 0.0)
+    dip_c = np.zeros((len(rows), V.shape[1])); dip_Z = np.zeros(len(rows))
+    if dip is not None:
+        p_ib, cov_b = dip
+        for r in range(len(rows)):
+            far = nonempty & ~selmask[r]
+            dip_Z[r] = p_ib[far].sum()
+            if np.isfinite(lse_far[r]) and dip_Z[r] > 0:
+                dip_c[r] = np.tensordot(p_ib[far], cov_b[far], axes=(0, 0)) @ qres[r] / dip_Z[r]
+        o_far = o_far + dip_c
     # 3. exact attention over the retrieved clusters' visible keys (full query)
     u = np.arange(N)
     vis = (u // Bs < b) if causal else np.ones(N, bool)
@@ -479,7 +577,7 @@ def _segment(Q, K, V, a_k, qbar_i, muh_ib, kah_ib, nuh_ib, rows, b, *, sigma, Bs
     L = _lse(lses, 1)
     wts = np.exp(lses - L[:, None])
     O = wts[:, 0:1] * o_far + wts[:, 1:2] * o_ret + wts[:, 2:3] * o_loc + wts[:, 3:4] * o_near
-    return dict(O=O, L=L, sel=sel_rows, bsel=bsel, near_logit=near_logit, o_near=o_near, lse_near=lse_near, sel_gap=gap, selmask=selmask, score=score, qp=qp, qres=qres,
+    return dict(O=O, L=L, sel=sel_rows, bsel=bsel, dip_c=dip_c, dip_Z=dip_Z, nonempty=nonempty, near_logit=near_logit, o_near=o_near, lse_near=lse_near, sel_gap=gap, selmask=selmask, score=score, qp=qp, qres=qres,
                 far_logit=far_logit, exact_logit=np.where(ret_mask | loc_mask, logit, -np.inf),
                 o_far=o_far, lse_far=lse_far, o_ret=o_ret, lse_ret=lse_ret,
                 o_loc=o_loc, lse_loc=lse_loc)
@@ -500,14 +598,16 @@ def forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, 
     """MuSe attention for one head.  Returns a dict with O [N,Dv], LSE [N], sel [N,m] and the
     three component (o, lse) pairs.  `sel` forces the retrieved clusters (teacher forcing);
     `rows` restricts the computation to some queries (others are left zero / -inf / -1).
-    `dipole=1` adds the untilted pre-merged dipole correction to the far field; the paper
-    defines it without retrieval, so it requires m = 0.
+    `dipole=1` adds the untilted dipole correction to the far field, `dipole=2` the one whose shared
+    covariance is tilted at the mass-weighted mean query centroid (`a_q` gives the masses).  The paper
+    defines the pre-merged correction without retrieval (m = 0); with m > 0 each query's correction is
+    the merge over the clusters it did not retrieve (see _segment).
     `k2` > 0: two-level retrieval; per (query, selected cluster) only the k2 best earlier blocks
     are retrieved exactly (returned as bsel [N, m, k2], -1 padded; `bsel` forces them), the other
     earlier blocks of the selected clusters are approximated by their per-block summaries
     (`blocks` = block_summaries(...) may be passed in).  k2 = 0 retrieves every visible block."""
-    if dipole and m != 0:
-        raise ValueError("the dipole correction is defined for m = 0 (no retrieval)")
+    if dipole not in (0, 1, 2):
+        raise ValueError("dipole is 0 (off), 1 (untilted) or 2 (tilted at the mean query centroid)")
     if k2 < 0 or (k2 > 0 and dipole):
         raise ValueError("k2 must be >= 0 and is not combined with the dipole correction")
     Q = np.asarray(Q, np.float64); K = np.asarray(K, np.float64); V = np.asarray(V, np.float64)
@@ -521,7 +621,12 @@ def forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, 
     muh, kah, nuh = summ
     if k2 > 0 and causal and blocks is None:
         blocks = block_summaries(K, V, a_k, qbar, sigma, S, Ck)
-    cbar = merged_dipole(muh, untilted_covariances(K, V, a_k, S, Ck, causal)) if dipole else None
+    cbar = cov = pw = None
+    if dipole:
+        cov = (untilted_covariances(K, V, a_k, S, Ck, causal) if dipole == 1 else
+               tilted_covariances(K, V, a_k, S, Ck, mean_query_centroid(qbar, a_q), sigma, causal))
+        cbar = merged_dipole(muh, cov)
+        pw = dipole_weights(muh)
     out = dict(O=np.zeros((N, Dv)), LSE=np.full(N, -np.inf), sel=np.full((N, m), -1, np.int32),
                sel_gap=np.full(N, np.inf))
     for name in ("o_far", "o_ret", "o_loc", "o_near"):
@@ -534,9 +639,10 @@ def forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, 
         seg = _segment(Q, K, V, a_k, qbar[i], muh[b, i], kah[b, i], nuh[b, i], r, b,
                        sigma=sigma, Bs=Bs, m=m, causal=causal,
                        sel_rows=None if sel is None else sel[r], sel_mode=sel_mode,
-                       cbar_ib=None if cbar is None else cbar[b, i], k2=k2,
+                       cbar_ib=cbar[b, i] if (dipole and m == 0) else None, k2=k2,
                        blk_i=None if blocks is None else (blocks[0][:, i], blocks[1][:, i], blocks[2][:, i]),
-                       bsel_rows=None if bsel is None else bsel[r])
+                       bsel_rows=None if bsel is None else bsel[r],
+                       dip=(pw[b, i], cov[b]) if (dipole and m > 0) else None)
         out["O"][r], out["LSE"][r], out["sel"][r] = seg["O"], seg["L"], seg["sel"]
         out["sel_gap"][r] = seg["sel_gap"]
         for name in ("o_far", "lse_far", "o_ret", "lse_ret", "o_loc", "lse_loc", "o_near", "lse_near"):
@@ -545,17 +651,24 @@ def forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, 
             out["bsel"][r] = seg["bsel"]
     out["summ"] = summ
     out["cbar"] = cbar
+    out["cov"] = cov
     return out
 
 
 def backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None, sel_mode=0,
-             agg_grad=True, rows=None, k2=0, bsel=None):
+             agg_grad=True, rows=None, k2=0, bsel=None, dipole=0):
     """Gradients of sum(O * dO) w.r.t. Q, K, V with the assignments, the selections and the
     query centroids held constant (Appendix "Centroid Gradient Flow"; assignments and
     selections are discrete).  agg_grad=False also treats the tilted aggregation weights as
     constants (Appendix "Aggregation Weight Gradient Flow").  k2 > 0: two-level retrieval; the
     chosen blocks (`bsel`) are constants like the clusters, and the stand-in keys of the other
-    blocks pass their gradient on through the per-block summaries.  Returns (dQ, dK, dV, fwd)."""
+    blocks pass their gradient on through the per-block summaries.  `dipole` as in forward(): the
+    correction is differentiated through the residual, the shared covariances (to keys and values) and
+    the centroid weights p_ib(j) (to the log-masses, hence dropped with agg_grad=False, as is the
+    dependence of the dipole=2 tilt weights on the keys); the tilt point is a constant like qbar.
+    Returns (dQ, dK, dV, fwd)."""
+    if dipole not in (0, 1, 2) or (dipole and k2 > 0):
+        raise ValueError("dipole is 0, 1 or 2 and is not combined with k2 > 0")
     Q = np.asarray(Q, np.float64); K = np.asarray(K, np.float64); V = np.asarray(V, np.float64)
     dO = np.asarray(dO, np.float64); qbar = np.asarray(qbar, np.float64)
     N, D = Q.shape; Dv = V.shape[1]; Cq = qbar.shape[0]
@@ -569,6 +682,11 @@ def backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=N
         dmu_b = np.zeros_like(mu_b); dka_b = np.zeros_like(ka_b); dnu_b = np.zeros_like(nu_b)
     dQ = np.zeros((N, D)); dK = np.zeros((N, D)); dV = np.zeros((N, Dv))
     dmu = np.zeros_like(muh); dka = np.zeros_like(kah); dnu = np.zeros_like(nuh)
+    if dipole:
+        qstar = np.zeros(D) if dipole == 1 else mean_query_centroid(qbar, a_q)
+        cov = tilted_covariances(K, V, a_k, S, Ck, qstar, sigma, causal)
+        pw = dipole_weights(muh)
+        dcov = np.zeros_like(cov); dpw = np.zeros_like(pw)
     fwd = dict(O=np.zeros((N, Dv)), LSE=np.full(N, -np.inf), sel=np.full((N, m), -1, np.int32),
                sel_gap=np.full(N, np.inf))
     for b, i, r in _segments(a_q, N, S, causal, rows):
@@ -576,7 +694,8 @@ def backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=N
                        sigma=sigma, Bs=Bs, m=m, causal=causal,
                        sel_rows=None if sel is None else sel[r], sel_mode=sel_mode, k2=k2 if two_level else 0,
                        blk_i=(mu_b[:, i], ka_b[:, i], nu_b[:, i]) if two_level else None,
-                       bsel_rows=None if bsel is None else bsel[r])
+                       bsel_rows=None if bsel is None else bsel[r],
+                       dip=(pw[b, i], cov[b]) if dipole else None)
         fwd["O"][r], fwd["LSE"][r], fwd["sel"][r] = seg["O"], seg["L"], seg["sel"]
         fwd["sel_gap"][r] = seg["sel_gap"]
         L = seg["L"][:, None]
@@ -590,7 +709,8 @@ def backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=N
         dK += G.T @ seg["qp"]
         Pf = np.exp(seg["far_logit"] - L)                  # [n, Ck]
         dnu[b, i] += Pf.T @ g_out
-        Gf = Pf * (g_out @ nuh[b, i].T - delta)
+        # with the dipole every far cluster's value is nuh_j + c_t (c_t = the query's correction)
+        Gf = Pf * (g_out @ nuh[b, i].T + (g_out * seg["dip_c"]).sum(1, keepdims=True) - delta)
         dqp += Gf @ kah[b, i]                              # d score / d q = kah (qbar constant)
         dka[b, i] += Gf.T @ seg["qres"]
         dmu[b, i] += Gf.sum(0)
@@ -604,7 +724,24 @@ def backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=N
                 dqp += Gn @ ka_b[bp, i]
                 dka_b[bp, i] += Gn.T @ seg["qres"]
                 dmu_b[bp, i] += Gn.sum(0)
+        if dipole:
+            # c_t = M_t qres_t / Z_t,  M_t = sum_{j far} p(j) Cov_jb,  Z_t = sum_{j far} p(j)
+            w_far = np.exp(seg["lse_far"] - seg["L"])
+            for x in range(len(r)):
+                Z = seg["dip_Z"][x]
+                if not (np.isfinite(seg["lse_far"][x]) and Z > 0):
+                    continue
+                far = seg["nonempty"] & ~seg["selmask"][x]
+                dc = w_far[x] * g_out[x]
+                M = np.tensordot(pw[b, i][far], cov[b][far], axes=(0, 0))
+                dqp[x] += M.T @ dc / Z
+                dM = np.outer(dc, seg["qres"][x]) / Z
+                dcov[b][far] += pw[b, i][far][:, None, None] * dM
+                dpw[b, i][far] += (cov[b][far] * dM).sum((1, 2)) - (dc @ seg["dip_c"][x]) / Z
         dQ[r] = sigma * dqp
+    if dipole:
+        # softmax backward of the centroid weights into the accumulated log-masses
+        dmu += pw * (dpw - (pw * dpw).sum(2, keepdims=True))
     # through the accumulated summaries to the keys and values they were built from
     blk = np.arange(N) // Bs
     for b in range(S):
@@ -622,6 +759,23 @@ def backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=N
                           + dka[b, :, j] @ K[mem].T - (dka[b, :, j] * kah[b, :, j]).sum(1)[:, None]
                           + dnu[b, :, j] @ V[mem].T - (dnu[b, :, j] * nuh[b, :, j]).sum(1)[:, None])
                 dK[mem] += sigma * (dl.T @ qbar)
+    if dipole:
+        # through the shared covariances: Cov = sum_u w_u (v_u - vm)(k_u - km)^T over the visible members
+        for b in range(S):
+            for j in range(Ck):
+                vis = (blk < b) if causal else np.ones(N, bool)
+                mem = np.nonzero(vis & (a_k == j))[0]
+                if mem.size == 0:
+                    continue
+                l = sigma * (K[mem] @ qstar)
+                w = np.exp(l - l.max()); w /= w.sum()
+                kc = K[mem] - w @ K[mem]; vc = V[mem] - w @ V[mem]
+                G = dcov[b, j]
+                dV[mem] += w[:, None] * (kc @ G.T)
+                dK[mem] += w[:, None] * (vc @ G)
+                if agg_grad and dipole == 2:
+                    dl = w * (((vc @ G) * kc).sum(1) - (G * cov[b, j]).sum())
+                    dK[mem] += sigma * dl[:, None] * qstar[None, :]
     if two_level:
         # ... and through the per-block summaries to the keys and values of their own bucket
         for bp in range(S):
@@ -667,7 +821,7 @@ def layer_forward(Q, K, V, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=
 
 
 def layer_backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True, sel=None,
-                   sel_mode=0, agg_grad=True, head_map=None, k2=0, bsel=None):
+                   sel_mode=0, agg_grad=True, head_map=None, k2=0, bsel=None, dipole=0):
     """dK, dV of a kv head are the sums over the query heads that share it."""
     B, Hq, N, D = Q.shape
     Hkv = K.shape[1]
@@ -679,7 +833,8 @@ def layer_backward(Q, K, V, dO, a_q, a_k, qbar, *, sigma, S, Ck, m, causal=True,
             q, k, v, _ = backward(Q[b, h], K[b, g], V[b, g], dO[b, h], a_q[b, h], a_k[b, g],
                                   qbar[b, h], sigma=sigma, S=S, Ck=Ck, m=m, causal=causal,
                                   sel=None if sel is None else sel[b, h], sel_mode=sel_mode,
-                                  agg_grad=agg_grad, k2=k2, bsel=None if bsel is None else bsel[b, h])
+                                  agg_grad=agg_grad, k2=k2, bsel=None if bsel is None else bsel[b, h],
+                                  dipole=dipole)
             dQ[b, h] = q
             dK[b, g] += k
             dV[b, g] += v
