@@ -62,7 +62,7 @@ typedef struct CUstream_st* cudaStream_t;
 
 enum { MUSE_BF16 = 0, MUSE_F32 = 1 };
 enum { MUSE_SEL_PER_QUERY = 0, MUSE_SEL_PER_QCLUSTER = 1 };
-enum { MUSE_INIT_INDICES = 0, MUSE_INIT_STRIDED = 1, MUSE_INIT_CENTRES = 2 };
+enum { MUSE_INIT_INDICES = 0, MUSE_INIT_STRIDED = 1, MUSE_INIT_CENTRES = 2, MUSE_INIT_KMEANSPP = 3 };
 /* Device status word (see "Device status" below): first code reported by a kernel of the call. */
 enum {
   MUSE_STATUS_OK = 0,
@@ -96,7 +96,7 @@ typedef struct muse_params {
   float   softmax_scale;        /* sigma; <= 0 -> 1/sqrt(D)                                        */
   int32_t kmeans_iters;         /* T Lloyd iterations before the final assignment (>= 0)           */
   int32_t init_mode;            /* MUSE_INIT_*                                                     */
-  uint64_t seed;                /* used by MUSE_INIT_STRIDED                                       */
+  uint64_t seed;                /* used by MUSE_INIT_STRIDED and MUSE_INIT_KMEANSPP                */
   int32_t sel_mode;             /* MUSE_SEL_*: rank clusters by the Eq. 6 score per query, or by
                                    the accumulated log-mass per (query cluster, block)            */
   int32_t dipole;               /* 0 off; 1: untilted, pre-merged dipole correction of the far field
@@ -143,6 +143,7 @@ MUSE_API int muse_summaries_layout(const muse_params_t* p, size_t off[9]);
  *   assign_q/k  out  [B,Hq,N] / [B,Hkv,N] cluster of every query / key
  *   qbar, kcent out  [B,Hq,Cq,D] / [B,Hkv,Ck,D] fp32 centres used by the final assignment;
  *                    with MUSE_INIT_CENTRES they are also the input start centres.
+ *   MUSE_INIT_KMEANSPP: the start points are drawn on the GPU by muse_kmeanspp_init.
  * Either side may be skipped by passing its Q/K pointer as NULL. */
 MUSE_API int muse_cluster(const muse_params_t* p, const void* Q, const void* K,
                  const int32_t* init_q, const int32_t* init_k,
@@ -229,6 +230,18 @@ MUSE_API int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K,
                   const int32_t* off_k, const int32_t* perm_k, const void* summaries,
                   const int32_t* sel, const int32_t* bsel, void* dQ, void* dK, void* dV,
                   void* ws, size_t ws_bytes, cudaStream_t stream);
+
+/* Seeded k-means++ start points, drawn on the GPU (the paper starts from a strided sample, Appendix
+ * "Centroid Computation" step 1; this is the usual better-spread alternative for the Lloyd iterations).
+ * Per head of side 0 (queries X = [B,Hq,N,D], C_q points) or 1 (keys [B,Hkv,N,D], C_k points): the first
+ * start point is position 0 of the seeded shuffle; draw c = 1 .. C-1 takes vector t with probability
+ * d2_t / sum d2, d2 = squared distance (fp32) to the nearest start point so far.  The draw is an exponential
+ * race, reproducible from p->seed alone: u_t = ((h >> 41) + 1/2) / 2^23 with h = splitmix64(splitmix64(seed
+ * ^ stream << 32 ^ 0xA5 << 56 ^ c) ^ t), stream = 2 * head + side; the largest d2_t / -log(u_t) wins, the
+ * lower index on ties.  idx_out [problems, C] int32 (DEVICE, out).  ws: muse_workspace_bytes out[0].
+ * Errors as for muse_cluster. */
+MUSE_API int muse_kmeanspp_init(const muse_params_t* p, const void* X, int side, int32_t* idx_out,
+                                void* ws, size_t ws_bytes, cudaStream_t stream);
 
 /* The paper's own clustering (Appendix "Clustering Details").  An alternative to muse_cluster with the
  * same outputs; the rest of the path does not care which produced them.

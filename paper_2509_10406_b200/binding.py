@@ -19,10 +19,11 @@ LIB_PATH = os.path.join(_HERE, os.path.basename(os.environ.get("MUSE_LIBRARY", "
 
 MUSE_BF16, MUSE_F32 = 0, 1
 MUSE_SEL_PER_QUERY, MUSE_SEL_PER_QCLUSTER = 0, 1
-MUSE_INIT_INDICES, MUSE_INIT_STRIDED, MUSE_INIT_CENTRES = 0, 1, 2
+MUSE_INIT_INDICES, MUSE_INIT_STRIDED, MUSE_INIT_CENTRES, MUSE_INIT_KMEANSPP = 0, 1, 2, 3
 
 EXPORTS = ("muse_workspace_bytes", "muse_summaries_layout", "muse_cluster", "muse_summarize",
            "muse_attn_fwd", "muse_attn_bwd", "muse_stream_workspace_bytes", "muse_stream_kmeans", "muse_balanced_assign",
+           "muse_kmeanspp_init",
            "muse_cluster_streaming", "muse_cluster_noalloc", "muse_cluster_noalloc_max_bytes",
            "muse_cluster_noalloc_status_copy", "muse_status_copy", "muse_test_force_paths",
            "muse_test_wait_timeout", "muse_debug_report", "muse_profile", "muse_profile_report", "muse_strerror")
@@ -207,6 +208,11 @@ def muse_stream_kmeans(p, X, side, totals, counts, centres, ws, beta=0.9, first_
     _check(lib().muse_stream_kmeans(ctypes.byref(p), _ptr(X), int(side), float(beta), int(first_batch), int(n_batches),
                                     _ptr(totals), _ptr(counts), _ptr(centres), _ptr(assign_stream), _ptr(ws),
                                     ws.numel() * ws.element_size(), _stream()), "muse_stream_kmeans")
+
+
+def muse_kmeanspp_init(p, X, side, idx_out, ws):
+    _check(lib().muse_kmeanspp_init(ctypes.byref(p), _ptr(X), int(side), _ptr(idx_out), _ptr(ws),
+                                    ws.numel() * ws.element_size(), _stream()), "muse_kmeanspp_init")
 
 
 def muse_balanced_assign(p, X, side, centres, assign, ws, cap_factor=4.0):

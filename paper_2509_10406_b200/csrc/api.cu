@@ -33,7 +33,7 @@ int resolve(const muse_params_t* p, Dims* d) {
   if (p->Cq < 1 || p->Ck < 1 || p->m < 0 || p->m > p->Ck) return MUSE_ERR_INVALID_ARG;
   if (p->Cq > p->N || p->Ck > p->N) return MUSE_ERR_INVALID_ARG;
   if (p->dtype != MUSE_BF16 && p->dtype != MUSE_F32) return MUSE_ERR_INVALID_ARG;
-  if (p->kmeans_iters < 0 || p->init_mode < 0 || p->init_mode > 2) return MUSE_ERR_INVALID_ARG;
+  if (p->kmeans_iters < 0 || p->init_mode < 0 || p->init_mode > 3) return MUSE_ERR_INVALID_ARG;
   if (p->sel_mode != MUSE_SEL_PER_QUERY && p->sel_mode != MUSE_SEL_PER_QCLUSTER) return MUSE_ERR_INVALID_ARG;
   if (p->n_blocks < 0 || p->k2 < 0) return MUSE_ERR_INVALID_ARG;
   if (p->D != 64 && p->D != 128) return MUSE_ERR_UNSUPPORTED;
@@ -200,6 +200,24 @@ int muse_stream_workspace_bytes(const muse_params_t* p, size_t* bytes) {
   const size_t tot = std::max(pq * d.Cq, pk * d.Ck);
   *bytes = up256(bal) + up256(tot * d.D * sizeof(float)) + up256(tot * sizeof(float));
   return MUSE_OK;
+}
+
+int muse_kmeanspp_init(const muse_params_t* p, const void* X, int side, int32_t* idx_out, void* ws, size_t ws_bytes,
+                       cudaStream_t stream) {
+  Dims d;
+  int rc = resolve(p, &d);
+  if (rc != MUSE_OK) return rc;
+  if (!X || !idx_out || !ws || (side != 0 && side != 1)) return MUSE_ERR_INVALID_ARG;
+  if (!aligned16(X) || !aligned16(ws)) return MUSE_ERR_INVALID_ARG;
+  const int problems = side == 0 ? d.B * d.Hq : d.B * d.Hkv, C = side == 0 ? d.Cq : d.Ck;
+  if (ws_bytes < up256(kStatusWords * sizeof(int32_t)) + up256((size_t)problems * d.N * sizeof(float))) return MUSE_ERR_WORKSPACE;
+  if (clear_status(ws, stream) != MUSE_OK) return MUSE_ERR_CUDA;
+  Arena ar(ws);
+  ar.take<int32_t>(kStatusWords);
+  float* mind2 = ar.take<float>((size_t)problems * d.N);
+  rc = kmeanspp(p->dtype, X, problems, d.N, d.D, C, side, p->seed, mind2, idx_out, stream);
+  prof_mark(nullptr, stream);
+  return rc;
 }
 
 int muse_stream_kmeans(const muse_params_t* p, const void* X, int side, float beta, int first_batch, int n_batches,

@@ -394,6 +394,15 @@ static int lloyd_t(const Dims& d, const T* X, int problems, int C, int kind, con
   __nv_bfloat16* chi = ar.take<__nv_bfloat16>((size_t)problems * C * D);
   __nv_bfloat16* clo = ar.take<__nv_bfloat16>((size_t)problems * C * D);
   constexpr bool kTensor = sizeof(T) == 2;     // bf16 inputs: distances on the tensor cores
+  if (init_mode == MUSE_INIT_KMEANSPP) {
+    // the draws borrow two arrays that the iterations only fill later: perm as the running minimum distance
+    // [problems, N] fp32, off (at least C + 1 words per problem) as the drawn indices [problems, C]
+    int rc = kmeanspp(sizeof(T) == 2 ? MUSE_BF16 : MUSE_F32, X, problems, d.N, D, C, kind, seed, reinterpret_cast<float*>(perm),
+                      off, st);
+    if (rc != MUSE_OK) return rc;
+    init_idx = off;
+    init_mode = MUSE_INIT_INDICES;
+  }
   if (init_mode != MUSE_INIT_CENTRES) {
     prof_mark("k_init_centres", st);
     k_init_centres<T><<<dim3(C, problems), 32, 0, st>>>(X, d.N, D, C, init_idx, init_mode, seed, kind, centres);

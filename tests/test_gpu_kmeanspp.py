@@ -1,0 +1,98 @@
+"""GPU parity of the seeded k-means++ start against the fp64 oracle.
+
+The draws form a chain (each depends on all earlier ones), so the gate is teacher-forced per draw: from the GPU's own
+earlier start points the oracle recomputes the squared distances and the race keys of draw c in fp64; the GPU's pick
+must be the oracle's, or a near-tie of it (its oracle key within 1e-5 relative of the largest)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import muse_oracle as orc
+from paper_2509_10406_b200 import workloads as wl
+from tests.gpu_util import Case, to_dev, to_np, kernels_launched
+from tests.test_gpu_cluster import CASES
+
+pytestmark = pytest.mark.gpu
+
+PP_CASES = dict(CASES)
+PP_CASES["ragged_cluster8"] = wl.WORKLOADS["headline"].with_(name="pp8", B=1, Hq=2, Hkv=1, N=16000, Cq=20, Ck=48, m=4, S=4,
+                                                           components=64)
+
+
+def _mb():
+    from paper_2509_10406_b200 import binding as mb
+    return mb
+
+
+@pytest.mark.parametrize("name", ["tiny", "gqa_bf16", "d128", "ragged_cluster8"])
+def test_kmeanspp_draws_teacher_forced(name):
+    mb = _mb()
+    c = Case(PP_CASES[name], gain=1.0, cluster=False)
+    w = c.w
+    p = c.params(seed=w.seed)
+    ws = torch.zeros(mb.muse_workspace_bytes(p)[0], dtype=torch.uint8, device="cuda")
+    Q, K, _, _ = c.dev()
+    near = total = 0
+    for side, X, Xd, H, C in ((0, c.Q, Q, w.Hq, w.Cq), (1, c.K, K, w.Hkv, w.Ck)):
+        P = w.B * H
+        idx = torch.full((P, C), -1, dtype=torch.int32, device="cuda")
+        with kernels_launched() as rec:
+            mb.muse_kmeanspp_init(p, Xd, side, idx, ws)
+        assert rec.names == {"k_kmeanspp"}, rec.names
+        assert mb.muse_status(ws) == 0
+        got = to_np(idx)
+        Xf = X.reshape(P, w.N, w.D)
+        for pr in range(P):
+            stream = pr * 2 + side
+            assert got[pr, 0] == orc.feistel_permute(0, w.N, w.seed, stream)
+            assert len(set(got[pr].tolist())) == C and got[pr].min() >= 0 and got[pr].max() < w.N
+            d2 = ((Xf[pr] - Xf[pr][got[pr, 0]]) ** 2).sum(1)
+            for cc in range(1, C):
+                want, keys = orc.kmeanspp_step(d2, cc, w.seed, stream)
+                if got[pr, cc] != want:
+                    assert keys[got[pr, cc]] >= keys[want] * (1 - 1e-5), (name, side, pr, cc)
+                    near += 1
+                total += 1
+                d2 = np.minimum(d2, ((Xf[pr] - Xf[pr][got[pr, cc]]) ** 2).sum(1))
+    assert near <= 0.01 * total + 1
+    print(f"[{name}] near-tie differences {near} of {total}")
+
+
+def test_cluster_with_kmeanspp_start_equals_cluster_from_the_same_indices():
+    mb = _mb()
+    c = Case(CASES["gqa_bf16"], gain=1.0, cluster=False)
+    w = c.w
+    Q, K, _, _ = c.dev()
+    res = []
+    p1 = c.params(seed=11, init_mode=mb.MUSE_INIT_KMEANSPP)
+    ws = torch.zeros(mb.muse_workspace_bytes(p1)[0], dtype=torch.uint8, device="cuda")
+    iq = torch.zeros(w.B * w.Hq, w.Cq, dtype=torch.int32, device="cuda"); ik = torch.zeros(w.B * w.Hkv, w.Ck, dtype=torch.int32, device="cuda")
+    mb.muse_kmeanspp_init(p1, Q, 0, iq, ws); mb.muse_kmeanspp_init(p1, K, 1, ik, ws)
+    for p, a, b in ((p1, None, None), (c.params(seed=11, init_mode=mb.MUSE_INIT_INDICES), iq, ik)):
+        aq = torch.zeros(w.B, w.Hq, w.N, dtype=torch.int32, device="cuda"); ak = torch.zeros(w.B, w.Hkv, w.N, dtype=torch.int32, device="cuda")
+        qb = torch.zeros(w.B, w.Hq, w.Cq, w.D, device="cuda"); kc = torch.zeros(w.B, w.Hkv, w.Ck, w.D, device="cuda")
+        with kernels_launched() as rec:
+            mb.muse_cluster(p, Q, K, a, b, aq, ak, qb, kc, ws)
+        assert ("k_kmeanspp" in rec.names) == (a is None)
+        assert mb.muse_status(ws) == 0
+        res.append((to_np(aq), to_np(ak), to_np(qb), to_np(kc)))
+    for x, y in zip(*res):
+        np.testing.assert_array_equal(x, y)
+
+
+def test_kmeanspp_start_spreads_over_separated_blobs():
+    """Sixteen tight, well separated blobs and sixteen start points: the D^2 law puts one in every blob (the strided
+    start does not), so the clustering that follows recovers the blobs."""
+    mb = _mb()
+    rng = np.random.default_rng(3)
+    N, D, C = 4096, 64, 16
+    cen = 40.0 * rng.standard_normal((C, D))
+    lab = rng.integers(0, C, N)
+    X = (cen[lab] + 0.05 * rng.standard_normal((N, D))).astype(np.float32)
+    p = mb.make_params(B=1, Hq=1, Hkv=1, N=N, D=D, Cq=C, Ck=C, m=2, n_blocks=4, dtype="f32", kmeans_iters=0, seed=5)
+    ws = torch.zeros(mb.muse_workspace_bytes(p)[0], dtype=torch.uint8, device="cuda")
+    idx = torch.zeros(1, C, dtype=torch.int32, device="cuda")
+    mb.muse_kmeanspp_init(p, to_dev(X[None, None], "f32"), 0, idx, ws)
+    got = to_np(idx)[0]
+    assert sorted(lab[got].tolist()) == list(range(C))
+    np.testing.assert_array_equal(got, orc.kmeanspp_init(X.astype(np.float64), C, 5, 0))
