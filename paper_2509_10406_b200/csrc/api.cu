@@ -40,7 +40,6 @@ int resolve(const muse_params_t* p, Dims* d) {
   if (p->Hq > kMaxHeads || p->m > kMaxM || p->Cq > kMaxC || p->Ck > kMaxC) return MUSE_ERR_UNSUPPORTED;
   if (p->dipole != 0 && p->dipole != 1) return MUSE_ERR_INVALID_ARG;
   if (p->k2 > 8 || (p->k2 > 0 && p->dipole != 0)) return MUSE_ERR_UNSUPPORTED;
-  if (p->dipole != 0 && p->m != 0) return MUSE_ERR_UNSUPPORTED;      // the paper defines the dipole without retrieval
   int S = p->causal ? (p->n_blocks == 0 ? 8 : p->n_blocks) : 1;
   if (p->N % S != 0) return MUSE_ERR_INVALID_ARG;
   if ((long long)S * p->Cq > 32768 || (long long)S * p->Ck > 32768) return MUSE_ERR_UNSUPPORTED;

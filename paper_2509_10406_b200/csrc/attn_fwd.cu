@@ -548,7 +548,7 @@ __global__ void k_merge(Dims dm, const float* __restrict__ o_far, const float* _
 // ---------------------------------------------------------------------------------------------
 template <class T> constexpr bool kTensorT() { return sizeof(T) == 2; }
 
-struct FwdWs { int32_t *status, *off_q, *perm_q, *sort_scratch, *ret_scratch, *sel_tmp, *bsel_tmp; float *o_far, *lse_far, *o_loc, *lse_loc, *o_part, *l_part, *o_near, *lse_near; };
+struct FwdWs { int32_t *status, *off_q, *perm_q, *sort_scratch, *ret_scratch, *sel_tmp, *bsel_tmp; float *o_far, *lse_far, *o_loc, *lse_loc, *o_part, *l_part, *o_near, *lse_near, *csub; };
 
 static FwdWs fwd_ws(const Dims& d, Arena& ar) {
   FwdWs w;
@@ -570,6 +570,7 @@ static FwdWs fwd_ws(const Dims& d, Arena& ar) {
   w.bsel_tmp = ar.take<int32_t>(two_level ? pq * d.N * d.m * d.k2 : 0);
   w.o_near = ar.take<float>(two_level ? pq * d.N * d.D : 0);
   w.lse_near = ar.take<float>(two_level ? pq * d.N : 0);
+  w.csub = ar.take<float>(d.dipole && d.m > 0 && d.SB > 0 ? pq * d.N * d.D : 0);
   return w;
 }
 
@@ -619,10 +620,6 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
           d, Q, qbar, w.off_q, w.perm_q, summ_ptrs(L, base), sel_in, sel, w.o_far, w.lse_far);
       MUSE_LAUNCH_OK();
     }
-    if (d.dipole) {
-      rc = dipole_apply(d, dtype, Q, qbar, w.off_q, w.perm_q, base + L.cbar, w.lse_far, w.o_far, st);
-      if (rc != MUSE_OK) return rc;
-    }
     if (two_level) {
       // second level: the k2 best earlier blocks of every selected cluster, and the near field of the others
       if (block_select_q_supported(d, dtype) && !path_forced(kForceBlockSelectWarp))
@@ -631,10 +628,20 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
       rc = block_select(d, dtype, Q, w.off_q, w.perm_q, sel, summ_ptrs_blk(L, base), bsel_in, bsel, w.o_near, w.lse_near, st);
       if (rc != MUSE_OK) return rc;
     }
+    if (d.dipole && d.m == 0) {
+      rc = dipole_apply(d, dtype, Q, qbar, assign_q, w.off_q, w.perm_q, dipole_ptrs(L, base), w.lse_far, nullptr, nullptr, nullptr,
+                        nullptr, w.o_far, nullptr, nullptr, st);
+      if (rc != MUSE_OK) return rc;
+    }
     if (d.m > 0) {
       RetIndex ri;
       rc = build_ret_index(d, sel, bsel, w.ret_scratch, &ri, st);
       if (rc != MUSE_OK) return rc;
+      if (d.dipole) {
+        rc = dipole_apply(d, dtype, Q, qbar, assign_q, w.off_q, w.perm_q, dipole_ptrs(L, base), w.lse_far, sel, ri.goff, ri.pairs,
+                          w.csub, w.o_far, nullptr, nullptr, st);
+        if (rc != MUSE_OK) return rc;
+      }
       if (kTensor) {
         rc = ret_fwd_tc(d, Q, Kp, Vp, off_k, ri.goff, ri.pairs, w.o_part, w.l_part, w.status, st);
         if (rc != MUSE_OK) return rc;

@@ -22,7 +22,7 @@ struct Dims {
   int SB;       // stored summary planes: S-1 (causal) or 1
   int Bs;       // block size N / S
   int causal, sel_mode, agg_grad;
-  int dipole;   // 1: untilted pre-merged dipole correction of the far field (needs m == 0)
+  int dipole;   // 1: untilted dipole correction of the far field; with m > 0 restricted to the clusters a query did not retrieve
   int k2;       // spatial selection: 0 = every earlier block of a selected cluster is retrieved; > 0 = only the k2 best (causal only)
   float sigma;
   HeadMap hm;
@@ -174,12 +174,6 @@ size_t summarize_ws_bytes(const Dims& d, int dtype);
 // summary kernels load their centroid tiles from these by TMA instead of converting them per CTA
 int split_qbar(const Dims& d, const float* qbar, void* qhi, void* qlo, cudaStream_t st);
 
-// dipole correction (dipole.cu): construction at summary time, consumption after the far field
-size_t dipole_ws_bytes(const Dims& d, int dtype);
-int dipole_build(const Dims& d, int dtype, const void* Kp, const void* Vp, const int32_t* off_k, const float* mu,
-                 void* cbar, void* ws, int* status, cudaStream_t st);
-int dipole_apply(const Dims& d, int dtype, const void* Q, const float* qbar, const int32_t* off_q, const int32_t* perm_q,
-                 const void* cbar, const float* lse_far, float* o_far, cudaStream_t st);
 
 // Byte offsets inside the caller's summaries buffer.  Per entry (b, h, plane, i, j):
 //   mu   fp32  accumulated log-mass            beta fp32  mu - sigma qbar_i . kappa  (so that the
@@ -190,7 +184,7 @@ int dipole_apply(const Dims& d, int dtype, const void* Q, const float* qbar, con
 //   cbar (dipole only): merged dipole matrices [B,Hq,SB,Cq][D value dims][D key dims], fp32 or bf16
 //   blk (k2 > 0 only): a second set mu | beta | kappa (hi, lo) | nu with the same shapes holding the PER-BLOCK
 //              (pre-accumulation) summaries: plane s = the summary of the keys of block s alone
-struct SummLayout { size_t mu, beta, khi, klo, nu, Kp, Vp, cbar, blk, blk_beta, blk_khi, blk_klo, blk_nu, total; };
+struct SummLayout { size_t mu, beta, khi, klo, nu, Kp, Vp, cbar, cov, pw, zall, blk, blk_beta, blk_khi, blk_klo, blk_nu, total; };
 SummLayout summ_layout(const Dims& d, int dtype);
 
 struct SummPtrs { float* mu; float* beta; void* khi; void* klo; void* nu; };
@@ -198,10 +192,23 @@ inline SummPtrs summ_ptrs(const SummLayout& L, const void* base_) {
   char* b = (char*)base_;
   return SummPtrs{(float*)(b + L.mu), (float*)(b + L.beta), b + L.khi, b + L.klo, b + L.nu};
 }
+// dipole part of the summaries buffer: merged matrices, shared covariances, centroid weights and their sums
+struct DipolePtrs { void* cbar; void* cov; void* pw; float* zall; };
+inline DipolePtrs dipole_ptrs(const SummLayout& L, const void* base_) {
+  char* b = (char*)base_;
+  return DipolePtrs{b + L.cbar, b + L.cov, b + L.pw, (float*)(b + L.zall)};
+}
 inline SummPtrs summ_ptrs_blk(const SummLayout& L, const void* base_) {      // the per-block set (k2 > 0)
   char* b = (char*)base_;
   return SummPtrs{(float*)(b + L.blk), (float*)(b + L.blk_beta), b + L.blk_khi, b + L.blk_klo, b + L.blk_nu};
 }
+// dipole correction (dipole.cu): construction at summary time, consumption after the far field
+size_t dipole_fwd_ws_bytes(const Dims& d);
+int dipole_build(const Dims& d, int dtype, const void* Kp, const void* Vp, const int32_t* off_k, const float* mu,
+                 const DipolePtrs& dp, int* status, cudaStream_t st);
+int dipole_apply(const Dims& d, int dtype, const void* Q, const float* qbar, const int32_t* assign_q, const int32_t* off_q,
+                 const int32_t* perm_q, const DipolePtrs& dp, const float* lse_far, const int32_t* sel, const int32_t* goff,
+                 const int32_t* pairs, float* csub, float* o_far, float* corr, float* zq, cudaStream_t st);
 // ST = storage element type of kappa / nu (float or bf16); idx = element index (entry * D + d), d % 4 == 0
 template <class ST> __device__ __forceinline__ float4 ld_kappa4(const SummPtrs& s, size_t idx);
 template <> __device__ __forceinline__ float4 ld_kappa4<float>(const SummPtrs& s, size_t idx) { return ld4((const float*)s.khi + idx); }

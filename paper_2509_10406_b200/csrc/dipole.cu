@@ -6,13 +6,21 @@
 //   3. Cbar_ib = sum_j p_ib(j) Cov_0jb   -- one GEMM [Cq x Ck] x [Ck x D^2] per (head, plane);
 //      tcgen05 kernel in dipole_tc.cu, plain kernel here for fp32 mode and odd shapes
 //   4. o_far_t += Cbar_ib * sigma (q_t - qbar_i)   (value shift only; the mass is unchanged)
+// Next to retrieval (m > 0; Appendix "Compatibility with Retrieval") the clusters a query retrieved are attended
+// exactly, so their share leaves the merged matrix and the centroid weights are renormalised over the rest:
+//   c_t = (Cbar_ib qres_t - sum_{j in sel_t} p_ib(j) Cov_0jb qres_t) / (sum_j p_ib(j) - sum_{j in sel_t} p_ib(j)).
+// The subtraction only cancels cleanly if both sides hold the same numbers, so in this mode Cbar is kept in fp32
+// (the fp32 accumulation of exactly the stored, rounded weights and covariances) and the weight sums are taken
+// over the stored weights.  The retrieved clusters' terms are computed per (cluster, plane) group of the
+// retrieval's inverse index (one covariance in shared memory, its (query, slot) pairs streamed) and added
+// into a per-query row with floating-point atomics.
 #include "common.cuh"
 
 
 namespace muse {
 
 bool dipole_merge_tc_supported(const Dims& d, int dtype);
-int dipole_merge_tc(const Dims& d, const void* P, const void* cov, void* cbar, int* status, cudaStream_t st);
+int dipole_merge_tc(const Dims& d, const void* P, const void* cov, void* cbar, int out_f32, int* status, cudaStream_t st);
 
 // ---- 1. untilted accumulated covariance ------------------------------------------------------
 // One CTA per (key cluster j, kv head): walks the cluster's buckets in block order with running
@@ -87,7 +95,7 @@ k_dipole_cov(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const 
 
 // ---- 2. merge weights: one warp per (head, plane, query cluster) row of log-masses ---------------
 template <class ST>
-__global__ void k_dipole_weights(const float* __restrict__ mu, long long rows, int Ck, ST* __restrict__ P) {
+__global__ void k_dipole_weights(const float* __restrict__ mu, long long rows, int Ck, ST* __restrict__ P, float* __restrict__ zall) {
   const long long row = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   if (row >= rows) return;
@@ -100,15 +108,22 @@ __global__ void k_dipole_weights(const float* __restrict__ mu, long long rows, i
     for (int j = lane; j < Ck; j += 32) s += expf(mr[j] - mx);
   s = warp_sum(s);
   const float inv = s > 0.f ? 1.f / s : 0.f;
-  for (int j = lane; j < Ck; j += 32) P[row * Ck + j] = from_f<ST>(mx == -INFINITY ? 0.f : expf(mr[j] - mx) * inv);
+  float z = 0.f;
+  for (int j = lane; j < Ck; j += 32) {
+    const ST v = from_f<ST>(mx == -INFINITY ? 0.f : expf(mr[j] - mx) * inv);
+    P[row * Ck + j] = v;
+    z += to_f(v);
+  }
+  z = warp_sum(z);
+  if (lane == 0) zall[row] = z;                  // sum of the weights as stored (1 up to their rounding)
 }
 
 // ---- 3. merge, plain version: thread = one of 256 columns of the D*D axis, 16 query clusters ------
 constexpr int kMrgI = 16, kMrgJ = 64;
 
-template <class ST>
+template <class ST, class OT>
 __global__ void __launch_bounds__(256)
-k_dipole_merge(Dims dm, const ST* __restrict__ P, const ST* __restrict__ cov, ST* __restrict__ cbar) {
+k_dipole_merge(Dims dm, const ST* __restrict__ P, const ST* __restrict__ cov, OT* __restrict__ cbar) {
   __shared__ float ps[kMrgI][kMrgJ];
   const int DD = dm.D * dm.D;
   const int x = blockIdx.x * 256 + threadIdx.x, i0 = blockIdx.y * kMrgI;
@@ -135,40 +150,121 @@ k_dipole_merge(Dims dm, const ST* __restrict__ P, const ST* __restrict__ cov, ST
   }
 #pragma unroll
   for (int a = 0; a < kMrgI; ++a)
-    if (i0 + a < dm.Cq) cbar[((size_t)pp * dm.Cq + i0 + a) * DD + x] = from_f<ST>(acc[a]);
+    if (i0 + a < dm.Cq) cbar[((size_t)pp * dm.Cq + i0 + a) * DD + x] = from_f<OT>(acc[a]);
 }
 
-// ---- 4. consumption: one CTA per (query cluster, plane, head) segment ------------------------------
+// ---- 4a. the retrieved clusters' share (m > 0): one CTA per (key cluster j, plane, head) group of the inverse index ----
 constexpr int kApplyQ = 8;
 
-template <class T, class ST, int D>
-__global__ void __launch_bounds__(256)
-k_dipole_apply(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, const int32_t* __restrict__ off_q,
-               const int32_t* __restrict__ perm_q, const ST* __restrict__ cbar, const float* __restrict__ lse_far,
-               float* __restrict__ o_far) {
-  extern __shared__ float smd[];
-  float* Ct = smd;                              // [D key dims][D + 1]: transposed matrix, value dim fastest
-  float* qs = Ct + D * (D + 1);                 // [2 * kApplyQ][D] residuals
-  const int i = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z, tid = threadIdx.x;
-  const int blk = dm.causal ? pl + 1 : 0;
-  const int32_t* oq = off_q + (size_t)pq * (dm.S * dm.Cq + 1) + (size_t)blk * dm.Cq + i;
-  const int p0 = oq[0], p1 = oq[1];
-  if (p0 >= p1) return;
-  const ST* cb = cbar + (((size_t)pq * dm.SB + pl) * dm.Cq + i) * D * D;
+// Covariance (row-major [value dim][key dim]) into shared memory, transposed: Ct[key dim][value dim], pitch D + 1.
+template <class CT, int D>
+__device__ __forceinline__ void load_cov_t(const CT* __restrict__ cb, float* Ct, int tid) {
   for (int e = tid; e < D * D / 4; e += 256) {
     const int dv = e / (D / 4), c4 = (e % (D / 4)) * 4;
     const float4 v = ld4(cb + (size_t)dv * D + c4);
     Ct[(c4 + 0) * (D + 1) + dv] = v.x; Ct[(c4 + 1) * (D + 1) + dv] = v.y;
     Ct[(c4 + 2) * (D + 1) + dv] = v.z; Ct[(c4 + 3) * (D + 1) + dv] = v.w;
   }
+}
+
+template <class T, class ST, int D>
+__global__ void __launch_bounds__(256)
+k_dipole_sub(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, const int32_t* __restrict__ assign_q,
+             const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs, const ST* __restrict__ cov,
+             const ST* __restrict__ pw, float* __restrict__ csub) {
+  constexpr int G = 256 / D, R = G * kApplyQ;   // query groups working side by side, pairs per pass
+  extern __shared__ float smd[];
+  float* Ct = smd;
+  float* qs = Ct + D * (D + 1);                 // [R][D] residuals
+  __shared__ int t_s[R], i_s[R];
+  __shared__ float p_s[R];
+  const int j = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z, tid = threadIdx.x;
+  const int32_t* go = goff + (size_t)pq * (dm.SB * dm.Ck + 1) + (size_t)j * dm.SB + pl;
+  const int g0 = go[0], g1 = go[1];
+  if (g0 >= g1) return;
+  const int pk = (pq / dm.Hq) * dm.Hkv + dm.hm.g[pq % dm.Hq];
+  const int pc = dm.dipole == 2 ? pq : pk;      // the tilted covariance belongs to a query head
+  load_cov_t<ST, D>(cov + (((size_t)pc * dm.SB + pl) * dm.Ck + j) * D * D, Ct, tid);
+  const T* Qp = Q + (size_t)pq * dm.N * D;
+  const int32_t* aq = assign_q + (size_t)pq * dm.N;
+  const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
+  const ST* pwb = pw + ((size_t)pq * dm.SB + pl) * dm.Cq * dm.Ck;
+  const int grp = tid / D, dv = tid % D;
+  for (int r0 = g0; r0 < g1; r0 += R) {
+    __syncthreads();
+    if (tid < R) {
+      int t = -1, i = 0;
+      if (r0 + tid < g1) {
+        t = pr[r0 + tid] / dm.m;
+        if (!MUSE_IN_RANGE(t, dm.N)) t = -1;
+      }
+      if (t >= 0) { i = aq[t]; if (!MUSE_IN_RANGE(i, dm.Cq)) { t = -1; i = 0; } }
+      t_s[tid] = t; i_s[tid] = i;
+      p_s[tid] = t >= 0 ? to_f(pwb[(size_t)i * dm.Ck + j]) : 0.f;
+    }
+    __syncthreads();
+    for (int e = tid; e < R * D; e += 256) {
+      const int r = e / D, dk = e % D, t = t_s[r];
+      qs[e] = t >= 0 ? dm.sigma * (to_f(Qp[(size_t)t * D + dk]) - qbar[((size_t)pq * dm.Cq + i_s[r]) * D + dk]) : 0.f;
+    }
+    __syncthreads();
+    float acc[kApplyQ];
+#pragma unroll
+    for (int a = 0; a < kApplyQ; ++a) acc[a] = 0.f;
+    const float* qg = qs + grp * kApplyQ * D;
+    for (int dk = 0; dk < D; ++dk) {
+      const float c = Ct[dk * (D + 1) + dv];
+#pragma unroll
+      for (int a = 0; a < kApplyQ; ++a) acc[a] = fmaf(c, qg[a * D + dk], acc[a]);
+    }
+#pragma unroll
+    for (int a = 0; a < kApplyQ; ++a) {
+      const int r = grp * kApplyQ + a, t = t_s[r];
+      if (t >= 0) atomicAdd(&csub[((size_t)pq * dm.N + t) * D + dv], p_s[r] * acc[a]);
+    }
+  }
+}
+
+// ---- 4b. consumption: one CTA per (query cluster, plane, head) segment --------------------------------
+// m == 0: o_far += Cbar qres.  m > 0: o_far += (Cbar qres - csub) / Z with Z = the stored weights' sum minus the
+// retrieved clusters' weights; corr / zq (optional) receive the correction and Z for the backward pass.
+template <class T, class ST, class CT, int D>
+__global__ void __launch_bounds__(256)
+k_dipole_apply(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, const int32_t* __restrict__ off_q,
+               const int32_t* __restrict__ perm_q, const CT* __restrict__ cbar, const float* __restrict__ lse_far,
+               const int32_t* __restrict__ sel, const ST* __restrict__ pw, const float* __restrict__ zall,
+               const float* __restrict__ csub, float* __restrict__ o_far, float* __restrict__ corr, float* __restrict__ zq) {
+  constexpr int G = 256 / D, R = G * kApplyQ;
+  extern __shared__ float smd[];
+  float* Ct = smd;                              // [D key dims][D + 1]: transposed matrix, value dim fastest
+  float* qs = Ct + D * (D + 1);                 // [R][D] residuals
+  __shared__ float z_s[R];
+  const int i = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z, tid = threadIdx.x;
+  const int blk = dm.causal ? pl + 1 : 0;
+  const int32_t* oq = off_q + (size_t)pq * (dm.S * dm.Cq + 1) + (size_t)blk * dm.Cq + i;
+  const int p0 = oq[0], p1 = oq[1];
+  if (p0 >= p1) return;
+  load_cov_t<CT, D>(cbar + (((size_t)pq * dm.SB + pl) * dm.Cq + i) * D * D, Ct, tid);
   const float* qb = qbar + ((size_t)pq * dm.Cq + i) * D;
   const T* Qp = Q + (size_t)pq * dm.N * D;
   const int32_t* pm = perm_q + (size_t)pq * dm.N;
-  constexpr int G = 256 / D;                    // query groups working side by side (2 or 4)
+  const size_t row = ((size_t)pq * dm.SB + pl) * dm.Cq + i;
   const int grp = tid / D, dv = tid % D;
-  for (int r0 = p0; r0 < p1; r0 += G * kApplyQ) {
+  for (int r0 = p0; r0 < p1; r0 += R) {
     __syncthreads();
-    for (int e = tid; e < G * kApplyQ * D; e += 256) {
+    if (tid < R) {
+      float z = 1.f;
+      if (dm.m > 0 && r0 + tid < p1) {
+        const int t = pm[r0 + tid];
+        z = zall[row];
+        for (int s = 0; s < dm.m; ++s) {
+          const int jj = sel[((size_t)pq * dm.N + t) * dm.m + s];
+          if (jj >= 0 && MUSE_IN_RANGE(jj, dm.Ck)) z -= to_f(pw[row * dm.Ck + jj]);
+        }
+      }
+      z_s[tid] = z;
+    }
+    for (int e = tid; e < R * D; e += 256) {
       const int r = e / D, dk = e % D;
       qs[e] = r0 + r < p1 ? dm.sigma * (to_f(Qp[(size_t)pm[r0 + r] * D + dk]) - qb[dk]) : 0.f;
     }
@@ -187,74 +283,101 @@ k_dipole_apply(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar,
       const int r = r0 + grp * kApplyQ + a;
       if (r < p1) {
         const size_t t = (size_t)pq * dm.N + pm[r];
-        if (lse_far[t] != -INFINITY) o_far[t * D + dv] += acc[a];
+        const float z = z_s[grp * kApplyQ + a];
+        float c = 0.f;
+        if (lse_far[t] != -INFINITY && z > 1e-30f) c = dm.m > 0 ? (acc[a] - csub[t * D + dv]) / z : acc[a];
+        if (o_far) o_far[t * D + dv] += c;
+        if (corr) { corr[t * D + dv] = c; if (dv == 0) zq[t] = z; }
       }
     }
   }
 }
 
 // ---- host side ------------------------------------------------------------------------------------
-size_t dipole_ws_bytes(const Dims& d, int dtype) {
-  if (!d.dipole || d.SB == 0) return 0;
-  const size_t es = dtype == MUSE_F32 ? 4 : 2;
+// Scratch of the forward pass (and of the backward's recomputation): the retrieved clusters' rows.
+size_t dipole_fwd_ws_bytes(const Dims& d) {
+  if (!d.dipole || d.m == 0 || d.SB == 0) return 0;
   Arena ar(nullptr);
-  ar.take<char>((size_t)d.B * d.Hkv * d.SB * d.Ck * d.D * d.D * es);
-  ar.take<char>((size_t)d.B * d.Hq * d.SB * d.Cq * d.Ck * es);
+  ar.take<float>((size_t)d.B * d.Hq * d.N * d.D);
   return ar.used;
 }
 
 template <class T, class ST, int D>
 static int dipole_build_t(const Dims& d, int dtype, const T* Kp, const T* Vp, const int32_t* off_k, const float* mu,
-                          ST* cbar, void* ws, int* status, cudaStream_t st) {
-  Arena ar(ws);
-  ST* cov = ar.take<ST>((size_t)d.B * d.Hkv * d.SB * d.Ck * D * D);
-  ST* P = ar.take<ST>((size_t)d.B * d.Hq * d.SB * d.Cq * d.Ck);
+                          const DipolePtrs& dp, int* status, cudaStream_t st) {
+  ST* cov = (ST*)dp.cov; ST* P = (ST*)dp.pw;
   prof_mark("k_dipole_cov", st);
   k_dipole_cov<T, ST, D><<<dim3(d.Ck, d.B * d.Hkv), 256, 0, st>>>(d, Kp, Vp, off_k, cov);
   MUSE_LAUNCH_OK();
   const long long rows = (long long)d.B * d.Hq * d.SB * d.Cq;
   prof_mark("k_dipole_weights", st);
-  k_dipole_weights<ST><<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(mu, rows, d.Ck, P);
+  k_dipole_weights<ST><<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(mu, rows, d.Ck, P, dp.zall);
   MUSE_LAUNCH_OK();
+  const bool f32out = d.m > 0 && sizeof(ST) == 2;        // next to retrieval the merged matrices stay in fp32
   if (dipole_merge_tc_supported(d, dtype) && !path_forced(kForceDipoleSimt))
-    return dipole_merge_tc(d, P, cov, cbar, status, st);
+    return dipole_merge_tc(d, P, cov, dp.cbar, f32out ? 1 : 0, status, st);
   prof_mark("k_dipole_merge", st);
-  k_dipole_merge<ST><<<dim3(D * D / 256, cdiv(d.Cq, kMrgI), d.B * d.Hq * d.SB), 256, 0, st>>>(d, P, cov, cbar);
+  const dim3 grid(D * D / 256, cdiv(d.Cq, kMrgI), d.B * d.Hq * d.SB);
+  if (f32out) k_dipole_merge<ST, float><<<grid, 256, 0, st>>>(d, P, cov, (float*)dp.cbar);
+  else k_dipole_merge<ST, ST><<<grid, 256, 0, st>>>(d, P, cov, (ST*)dp.cbar);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }
 
 int dipole_build(const Dims& d, int dtype, const void* Kp, const void* Vp, const int32_t* off_k, const float* mu,
-                 void* cbar, void* ws, int* status, cudaStream_t st) {
+                 const DipolePtrs& dp, int* status, cudaStream_t st) {
   typedef __nv_bfloat16 bf;
   if (dtype == MUSE_F32) {
-    if (d.D == 64) return dipole_build_t<float, float, 64>(d, dtype, (const float*)Kp, (const float*)Vp, off_k, mu, (float*)cbar, ws, status, st);
-    return dipole_build_t<float, float, 128>(d, dtype, (const float*)Kp, (const float*)Vp, off_k, mu, (float*)cbar, ws, status, st);
+    if (d.D == 64) return dipole_build_t<float, float, 64>(d, dtype, (const float*)Kp, (const float*)Vp, off_k, mu, dp, status, st);
+    return dipole_build_t<float, float, 128>(d, dtype, (const float*)Kp, (const float*)Vp, off_k, mu, dp, status, st);
   }
-  if (d.D == 64) return dipole_build_t<bf, bf, 64>(d, dtype, (const bf*)Kp, (const bf*)Vp, off_k, mu, (bf*)cbar, ws, status, st);
-  return dipole_build_t<bf, bf, 128>(d, dtype, (const bf*)Kp, (const bf*)Vp, off_k, mu, (bf*)cbar, ws, status, st);
+  if (d.D == 64) return dipole_build_t<bf, bf, 64>(d, dtype, (const bf*)Kp, (const bf*)Vp, off_k, mu, dp, status, st);
+  return dipole_build_t<bf, bf, 128>(d, dtype, (const bf*)Kp, (const bf*)Vp, off_k, mu, dp, status, st);
 }
 
 template <class T, class ST, int D>
-static int dipole_apply_t(const Dims& d, const T* Q, const float* qbar, const int32_t* off_q, const int32_t* perm_q,
-                          const ST* cbar, const float* lse_far, float* o_far, cudaStream_t st) {
+static int dipole_apply_t(const Dims& d, const T* Q, const float* qbar, const int32_t* assign_q, const int32_t* off_q,
+                          const int32_t* perm_q, const DipolePtrs& dp, const float* lse_far, const int32_t* sel,
+                          const int32_t* goff, const int32_t* pairs, float* csub, float* o_far, float* corr, float* zq,
+                          cudaStream_t st) {
   const size_t smem = (size_t)(D * (D + 1) + (256 / D) * kApplyQ * D) * sizeof(float);
-  MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_apply<T, ST, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const dim3 grid(d.Cq, d.SB, d.B * d.Hq);
+  if (d.m > 0) {
+    MUSE_CUDA_OK(cudaMemsetAsync(csub, 0, (size_t)d.B * d.Hq * d.N * D * sizeof(float), st));
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_sub<T, ST, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    prof_mark("k_dipole_sub", st);
+    k_dipole_sub<T, ST, D><<<dim3(d.Ck, d.SB, d.B * d.Hq), 256, smem, st>>>(d, Q, qbar, assign_q, goff, pairs, (const ST*)dp.cov,
+                                                                            (const ST*)dp.pw, csub);
+    MUSE_LAUNCH_OK();
+    if (sizeof(ST) == 2) {
+      MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_apply<T, ST, float, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      prof_mark("k_dipole_apply", st);
+      k_dipole_apply<T, ST, float, D><<<grid, 256, smem, st>>>(d, Q, qbar, off_q, perm_q, (const float*)dp.cbar, lse_far, sel,
+                                                               (const ST*)dp.pw, dp.zall, csub, o_far, corr, zq);
+      MUSE_LAUNCH_OK();
+      return MUSE_OK;
+    }
+  }
+  MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_apply<T, ST, ST, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prof_mark("k_dipole_apply", st);
-  k_dipole_apply<T, ST, D><<<dim3(d.Cq, d.SB, d.B * d.Hq), 256, smem, st>>>(d, Q, qbar, off_q, perm_q, cbar, lse_far, o_far);
+  k_dipole_apply<T, ST, ST, D><<<grid, 256, smem, st>>>(d, Q, qbar, off_q, perm_q, (const ST*)dp.cbar, lse_far, sel, (const ST*)dp.pw,
+                                                        dp.zall, csub, o_far, corr, zq);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }
 
-int dipole_apply(const Dims& d, int dtype, const void* Q, const float* qbar, const int32_t* off_q, const int32_t* perm_q,
-                 const void* cbar, const float* lse_far, float* o_far, cudaStream_t st) {
+// o_far += correction (forward); corr / zq non-null: the correction and its weight sum are written out instead
+// (o_far may then be NULL).  sel, goff, pairs, csub are used with m > 0 only.
+int dipole_apply(const Dims& d, int dtype, const void* Q, const float* qbar, const int32_t* assign_q, const int32_t* off_q,
+                 const int32_t* perm_q, const DipolePtrs& dp, const float* lse_far, const int32_t* sel, const int32_t* goff,
+                 const int32_t* pairs, float* csub, float* o_far, float* corr, float* zq, cudaStream_t st) {
   typedef __nv_bfloat16 bf;
   if (dtype == MUSE_F32) {
-    if (d.D == 64) return dipole_apply_t<float, float, 64>(d, (const float*)Q, qbar, off_q, perm_q, (const float*)cbar, lse_far, o_far, st);
-    return dipole_apply_t<float, float, 128>(d, (const float*)Q, qbar, off_q, perm_q, (const float*)cbar, lse_far, o_far, st);
+    if (d.D == 64) return dipole_apply_t<float, float, 64>(d, (const float*)Q, qbar, assign_q, off_q, perm_q, dp, lse_far, sel, goff, pairs, csub, o_far, corr, zq, st);
+    return dipole_apply_t<float, float, 128>(d, (const float*)Q, qbar, assign_q, off_q, perm_q, dp, lse_far, sel, goff, pairs, csub, o_far, corr, zq, st);
   }
-  if (d.D == 64) return dipole_apply_t<bf, bf, 64>(d, (const bf*)Q, qbar, off_q, perm_q, (const bf*)cbar, lse_far, o_far, st);
-  return dipole_apply_t<bf, bf, 128>(d, (const bf*)Q, qbar, off_q, perm_q, (const bf*)cbar, lse_far, o_far, st);
+  if (d.D == 64) return dipole_apply_t<bf, bf, 64>(d, (const bf*)Q, qbar, assign_q, off_q, perm_q, dp, lse_far, sel, goff, pairs, csub, o_far, corr, zq, st);
+  return dipole_apply_t<bf, bf, 128>(d, (const bf*)Q, qbar, assign_q, off_q, perm_q, dp, lse_far, sel, goff, pairs, csub, o_far, corr, zq, st);
 }
 
 }  // namespace muse

@@ -23,9 +23,10 @@ constexpr int kDmCols = 256;                         // TMEM columns: half 0 at 
 
 struct DmBars { uint64_t full[kDmStages], empty[kDmStages], done; };
 
+template <class OT>
 __global__ void __launch_bounds__(128)
 k_dipole_merge_tc(Dims dm, const __grid_constant__ CUtensorMap tm_p, const __grid_constant__ CUtensorMap tm_cov,
-                  bf16* __restrict__ cbar, int* __restrict__ status) {
+                  OT* __restrict__ cbar, int* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ DmBars bars;
   __shared__ uint32_t tbase_s;
@@ -92,17 +93,21 @@ k_dipole_merge_tc(Dims dm, const __grid_constant__ CUtensorMap tm_p, const __gri
   // epilogue: thread = accumulator row (query cluster); all threads run the TMEM loads
   for (int hf = 0; hf < halves; ++hf) {
     const int i = i0 + hf * 128 + tid;
-    bf16* out = cbar + ((size_t)pp * dm.Cq + i) * DD + x0;
+    OT* out = cbar + ((size_t)pp * dm.Cq + i) * DD + x0;
 #pragma unroll
     for (int q = 0; q < kDmN / 32; ++q) {
       float v[32];
       tc::tmem_ld32(tbase + ((uint32_t)(warp * 32) << 16) + hf * kDmN + 32 * q, v);
-      if (ok && i < dm.Cq) {
+      if (ok && i < dm.Cq && sizeof(OT) == 4) {
+#pragma unroll
+        for (int c = 0; c < 32; c += 4)
+          *reinterpret_cast<float4*>((float*)out + 32 * q + c) = make_float4(v[c], v[c + 1], v[c + 2], v[c + 3]);
+      } else if (ok && i < dm.Cq) {
 #pragma unroll
         for (int c = 0; c < 32; c += 8) {
           __nv_bfloat162 w0 = __floats2bfloat162_rn(v[c], v[c + 1]), w1 = __floats2bfloat162_rn(v[c + 2], v[c + 3]);
           __nv_bfloat162 w2 = __floats2bfloat162_rn(v[c + 4], v[c + 5]), w3 = __floats2bfloat162_rn(v[c + 6], v[c + 7]);
-          *reinterpret_cast<uint4*>(out + 32 * q + c) = make_uint4(*reinterpret_cast<uint32_t*>(&w0), *reinterpret_cast<uint32_t*>(&w1),
+          *reinterpret_cast<uint4*>((bf16*)out + 32 * q + c) = make_uint4(*reinterpret_cast<uint32_t*>(&w0), *reinterpret_cast<uint32_t*>(&w1),
                                                                     *reinterpret_cast<uint32_t*>(&w2), *reinterpret_cast<uint32_t*>(&w3));
         }
       }
@@ -120,15 +125,18 @@ bool dipole_merge_tc_supported(const Dims& d, int dtype) {
   return dtype == MUSE_BF16 && d.Ck % kDmK == 0 && (d.D * d.D) % kDmN == 0 && rows_p < (1ll << 31) && rows_c < (1ll << 31);
 }
 
-int dipole_merge_tc(const Dims& d, const void* P, const void* cov, void* cbar, int* status, cudaStream_t st) {
+int dipole_merge_tc(const Dims& d, const void* P, const void* cov, void* cbar, int out_f32, int* status, cudaStream_t st) {
   CUtensorMap tp, tcv;
   int rc = make_tmap_bf16_rows(&tp, P, (uint64_t)d.B * d.Hq * d.SB * d.Cq, d.Ck, 128);
   if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tcv, cov, (uint64_t)d.B * d.Hkv * d.SB * d.Ck, d.D * d.D, kDmK);
   if (rc != MUSE_OK) return rc;
   const size_t smem = (size_t)kDmStages * kDmStage + 1024;
-  MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_merge_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_merge_tc<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_merge_tc<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prof_mark("k_dipole_merge_tc", st);
-  k_dipole_merge_tc<<<dim3(d.D * d.D / kDmN, cdiv(d.Cq, 256), d.B * d.Hq * d.SB), 128, smem, st>>>(d, tp, tcv, (bf16*)cbar, status);
+  const dim3 grid(d.D * d.D / kDmN, cdiv(d.Cq, 256), d.B * d.Hq * d.SB);
+  if (out_f32) k_dipole_merge_tc<float><<<grid, 128, smem, st>>>(d, tp, tcv, (float*)cbar, status);
+  else k_dipole_merge_tc<bf16><<<grid, 128, smem, st>>>(d, tp, tcv, (bf16*)cbar, status);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }

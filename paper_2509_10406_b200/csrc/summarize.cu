@@ -23,7 +23,13 @@ SummLayout summ_layout(const Dims& d, int dtype) {
   L.Kp = up(L.nu + ent * d.D * es);
   L.Vp = up(L.Kp + (size_t)d.B * d.Hkv * d.N * d.D * es);
   L.cbar = up(L.Vp + (size_t)d.B * d.Hkv * d.N * d.D * es);
-  L.blk = up(L.cbar + (d.dipole ? (size_t)d.B * d.Hq * d.SB * d.Cq * d.D * d.D * es : 0));
+  // dipole: merged matrices (fp32 next to retrieval, where retrieved clusters are subtracted from them), then the
+  // shared covariances (per kv head; per query head when tilted), the centroid weights and the sums of the weights
+  const size_t ecb = d.m > 0 ? 4 : es, covh = d.dipole == 2 ? d.Hq : d.Hkv;
+  L.cov = up(L.cbar + (d.dipole ? (size_t)d.B * d.Hq * d.SB * d.Cq * d.D * d.D * ecb : 0));
+  L.pw = up(L.cov + (d.dipole ? (size_t)d.B * covh * d.SB * d.Ck * d.D * d.D * es : 0));
+  L.zall = up(L.pw + (d.dipole ? ent * es : 0));
+  L.blk = up(L.zall + (d.dipole ? (size_t)d.B * d.Hq * d.SB * d.Cq * sizeof(float) : 0));
   L.blk_beta = L.blk_khi = L.blk_klo = L.blk_nu = L.blk;
   L.total = L.blk;
   if (d.k2 > 0) {                                       // per-block summaries beside the accumulated ones
@@ -255,7 +261,7 @@ static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const i
   rc = summarize_planes<T, D>(d, dtype, Kp, Vp, off_k, qbar, summ_ptrs(L, base), 0, qsplit, status, st);
   if (rc == MUSE_OK && d.k2 > 0) rc = summarize_planes<T, D>(d, dtype, Kp, Vp, off_k, qbar, summ_ptrs_blk(L, base), 1, qsplit, status, st);
   if (rc != MUSE_OK || !d.dipole) return rc;
-  return dipole_build(d, dtype, Kp, Vp, off_k, summ_ptrs(L, base).mu, base + L.cbar, (char*)ws + ar.used, status, st);
+  return dipole_build(d, dtype, Kp, Vp, off_k, summ_ptrs(L, base).mu, dipole_ptrs(L, base), status, st);
 }
 
 template <class T, int D>
@@ -277,7 +283,7 @@ size_t summarize_ws_bytes(const Dims& d, int dtype) {
   ar.take<int32_t>(kStatusWords);
   ar.take<int32_t>((size_t)d.B * d.Hkv * sort_ws_elems(d.N, d.Ck * d.S));
   ar.take<__nv_bfloat16>(2 * (size_t)d.B * d.Hq * d.Cq * d.D);
-  return ar.used + dipole_ws_bytes(d, dtype);
+  return ar.used;
 }
 
 int summarize(const Dims& d, int dtype, const void* K, const void* V, const int32_t* assign_k,

@@ -1,6 +1,7 @@
-"""GPU parity for the dipole correction of the far field (untilted, pre-merged, m = 0): merged
-matrices and forward outputs against the fp64 oracle, teacher-forced clustering.  Tolerance:
-max-abs error relative to the oracle tensor's max-abs <= 1e-4 (fp32 mode), 2e-2 (bf16 mode)."""
+"""GPU parity for the dipole correction of the far field (untilted, pre-merged; alone with m = 0 and next to
+retrieval with m > 0, where the retrieved clusters leave the merged matrix): merged matrices and forward outputs
+against the fp64 oracle, teacher-forced clustering (and, with m > 0, the GPU's own selection handed to the oracle).
+Tolerance: max-abs error relative to the oracle tensor's max-abs <= 1e-4 (fp32 mode), 2e-2 (bf16 mode)."""
 import numpy as np
 import pytest
 import torch
@@ -18,13 +19,19 @@ DIPOLE_CASES = {
     "d128_bf16": (CASES["d128"].with_(m=0), True),                                      # tensor merge, ragged Cq = 24
     "d128_bf16_two_halves": (CASES["d128"].with_(m=0, Hq=1, Hkv=1, N=2048, Cq=160, Ck=64), True),
     "d128_f32_odd_ck": (CASES["d128"].with_(dtype="f32", m=0, Hq=1, Hkv=1, N=1000, Cq=8, Ck=24, S=4), True),
+    # next to retrieval
+    "tiny_f32_m2": (CASES["tiny"].with_(m=2), True),
+    "tiny_f32_m2_noncausal": (CASES["tiny"].with_(m=2), False),
+    "gqa_bf16_d64_m6": (CASES["gqa_bf16"].with_(B=1, Hq=4, Hkv=2, m=6), True),
+    "d128_bf16_m8": (CASES["d128"].with_(m=8), True),
+    "d128_f32_odd_ck_m5": (CASES["d128"].with_(dtype="f32", m=5, Hq=1, Hkv=1, N=1000, Cq=8, Ck=24, S=4), True),
 }
 
 
 def _cbar(mb, p, buf):
     off = mb.muse_summaries_layout(p)
     n = p.B * p.Hq * p.SB * p.Cq * p.D * p.D
-    if p.dtype == mb.MUSE_F32:
+    if p.dtype == mb.MUSE_F32 or p.m > 0:
         t = buf.summaries[off[7]:off[7] + 4 * n].view(torch.float32)
     else:
         t = buf.summaries[off[7]:off[7] + 2 * n].view(torch.bfloat16).float()
@@ -46,14 +53,14 @@ def test_dipole_forward_matches_oracle(name, gain):
     mb.muse_attn_fwd(p, Q, K, V, a_q, qb, buf.off_k, buf.perm_k, buf.summaries, None, buf.O, buf.LSE, buf.sel, buf.ws)
     torch.cuda.synchronize()
     assert int(buf.ws[:4].view(torch.int32)[0]) == 0
-    O, L, cb = to_np(buf.O), to_np(buf.LSE), _cbar(mb, p, buf)
+    O, L, cb, sel = to_np(buf.O), to_np(buf.LSE), _cbar(mb, p, buf), to_np(buf.sel)
     t = tol(w.dtype)
     S = w.S if causal else 1
     moved = 0.0
     for b in range(w.B):
         for h in range(w.Hq):
             g = c.hm[h]
-            kw = dict(sigma=c.sigma, S=w.S, Ck=w.Ck, m=0, causal=causal)
+            kw = dict(sigma=c.sigma, S=w.S, Ck=w.Ck, m=w.m, causal=causal, sel=sel[b, h] if w.m > 0 else None)
             f1 = orc.forward(c.Q[b, h], c.K[b, g], c.V[b, g], c.a_q[b, h], c.a_k[b, g], qbar32[b, h].astype(np.float64), dipole=1, **kw)
             f0 = orc.forward(c.Q[b, h], c.K[b, g], c.V[b, g], c.a_q[b, h], c.a_k[b, g], qbar32[b, h].astype(np.float64),
                              summ=f1["summ"], **kw)
@@ -75,9 +82,11 @@ def test_dipole_argument_rules():
     from paper_2509_10406_b200 import binding as mb
     w = CASES["tiny"]
     with pytest.raises(mb.MuseError):
-        mb.muse_workspace_bytes(mb.make_params(B=1, Hq=1, Hkv=1, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=2, dipole=1))
+        mb.muse_workspace_bytes(mb.make_params(B=1, Hq=1, Hkv=1, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=2, dipole=1, k2=1))
+    with pytest.raises(mb.MuseError):
+        mb.muse_workspace_bytes(mb.make_params(B=1, Hq=1, Hkv=1, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=2, dipole=3))
     p0 = mb.make_params(B=1, Hq=1, Hkv=1, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=0, dtype="f32")
     p1 = mb.make_params(B=1, Hq=1, Hkv=1, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=0, dtype="f32", dipole=1)
     s0, s1 = mb.muse_workspace_bytes(p0), mb.muse_workspace_bytes(p1)
-    assert s1[4] >= s0[4] + 7 * w.Cq * w.D * w.D * 4 and s1[1] > s0[1]
+    assert s1[4] >= s0[4] + 7 * (w.Cq + w.Ck) * w.D * w.D * 4
     assert mb.muse_summaries_layout(p0)[7] == s0[4]
