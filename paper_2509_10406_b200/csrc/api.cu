@@ -330,7 +330,7 @@ int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K, const vo
   int rc = resolve(p, &d);
   if (rc != MUSE_OK) return rc;
   if (!Q || !K || !V || !O || !LSE || !dO || !assign_q || !qbar || !off_k || !perm_k || !dQ || !dK || !dV || !ws) return MUSE_ERR_INVALID_ARG;
-  if (d.dipole) return MUSE_ERR_UNSUPPORTED;       // no backward through the dipole correction
+  if (d.dipole && !dipole_bwd_supported(d)) return MUSE_ERR_UNSUPPORTED;
   if (d.m > 0 && d.SB > 0 && sel == nullptr) return MUSE_ERR_INVALID_ARG;
   if (d.k2 > 0 && d.m > 0 && d.SB > 0 && bsel == nullptr) return MUSE_ERR_INVALID_ARG;   // the forward pass's chosen blocks
   if (!aligned16(Q) || !aligned16(K) || !aligned16(V) || !aligned16(O) || !aligned16(dO) || !aligned16(qbar) ||

@@ -676,6 +676,7 @@ struct BwdWs {
   __nv_bfloat16* qsplit;
   float *delta, *dQacc, *dq_part, *dK_orig, *dV_orig, *dK_perm, *dV_perm, *dkappa, *dnu, *dS;
   float *dkappa_b, *dnu_b, *dS_b;           // gradients of the per-block summaries (two-level retrieval), fp32
+  DipoleBwdWs dip;                          // dipole correction
 };
 
 static BwdWs bwd_ws(const Dims& d, Arena& ar) {
@@ -703,6 +704,7 @@ static BwdWs bwd_ws(const Dims& d, Arena& ar) {
     w.dnu_b = ar.take<float>(ent * d.D);
     w.dS_b = ar.take<float>(ent);
   }
+  w.dip = dipole_bwd_ws(d, ar);
   return w;
 }
 
@@ -753,8 +755,8 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
   if (d.SB > 0) {
     int rc = bucket_sort(0, assign_q, pq, d.N, d.Cq, d.S, d.Bs, 0, w.off_q, w.perm_q, w.sort_scratch, st);
     if (rc != MUSE_OK) return rc;
+    RetIndex ri = {};
     if (d.m > 0) {
-      RetIndex ri;
       rc = build_ret_index(d, sel, bsel, w.ret_scratch, &ri, st);
       if (rc != MUSE_OK) return rc;
       if (kTensor) {
@@ -769,18 +771,36 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
       }
       use_ret = 1;
     }
+    const float* delta_far = w.delta;
+    if (d.dipole) {
+      // the forward's far log-sum-exp, correction and weight sums again; then everything of the dipole's backward that
+      // does not need the far-field backward's output
+      const DipolePtrs dp = dipole_ptrs(L, base);
+      rc = far_fwd_again(d, dtype, Q, qbar, w.off_q, w.perm_q, sp, sel, w.dip.sel_tmp, w.dip.xq, w.dip.lse_far, w.status, st);
+      if (rc != MUSE_OK) return rc;
+      rc = dipole_apply(d, dtype, Q, qbar, assign_q, w.off_q, w.perm_q, dp, w.dip.lse_far, sel, ri.goff, ri.pairs, w.dip.csub, nullptr,
+                        w.dip.corr, w.dip.zq, st);
+      if (rc != MUSE_OK) return rc;
+      rc = dipole_bwd_pre(d, dtype, Q, dO, qbar, LSE, w.delta, assign_q, w.off_q, w.perm_q, dp, ri.goff, ri.pairs, w.dip, w.dQacc, st);
+      if (rc != MUSE_OK) return rc;
+      delta_far = w.dip.delta_far;
+    }
     const bool far_tc = far_bwd_tc_supported(d, dtype) && !path_forced(kForceFarSimt);
     const size_t fsm = (size_t)(4 * kTile * (D + 4) + kTile * kLDP) * sizeof(float) + (size_t)kTile * cdiv(d.Ck, 32) * sizeof(uint32_t);
     const bool summ_tc = far_tc && summ_bwd_tc_supported(d, dtype) && !path_forced(kForceSummBwdSimt);
     if (far_tc) {
-      rc = far_bwd_tc(d, sp, Q, dO, qbar, LSE, w.delta, w.off_q, w.perm_q, sel, w.dQacc, w.dkappa, w.dnu, w.dS, summ_tc ? 1 : 0, w.status, st);
+      rc = far_bwd_tc(d, sp, Q, dO, qbar, LSE, delta_far, w.off_q, w.perm_q, sel, w.dQacc, w.dkappa, w.dnu, w.dS, summ_tc ? 1 : 0, w.status, st);
       if (rc != MUSE_OK) return rc;
     } else {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fsm));
     prof_mark("k_far_bwd", st);
-    k_far_bwd<T, D><<<dim3(d.Cq, d.SB, pq), kFlashThreads, fsm, st>>>(d, Q, dO, qbar, LSE, w.delta, w.off_q, w.perm_q, sel, sp,
+    k_far_bwd<T, D><<<dim3(d.Cq, d.SB, pq), kFlashThreads, fsm, st>>>(d, Q, dO, qbar, LSE, delta_far, w.off_q, w.perm_q, sel, sp,
                                                                     w.dQacc, w.dkappa, w.dnu, w.dS);
     MUSE_LAUNCH_OK();
+    }
+    if (d.dipole) {
+      rc = dipole_bwd_dmu(d, dtype, dipole_ptrs(L, base), w.dip, w.dS, summ_tc ? 1 : 0, st);
+      if (rc != MUSE_OK) return rc;
     }
     const size_t ssm = (size_t)(5 * kTile * (D + 4) + kTile * kLDP) * sizeof(float);
     if (summ_tc) {
@@ -799,6 +819,10 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
                                                                         w.dK_perm, w.dV_perm, 0);
     }
     MUSE_LAUNCH_OK();
+    if (d.dipole) {
+      rc = dipole_bwd_keys(d, dtype, Kp, Vp, off_k, w.dip, w.dK_perm, w.dV_perm, st);
+      if (rc != MUSE_OK) return rc;
+    }
   }
   if (d.k2 > 0 && d.m > 0 && d.SB > 0) {
     // two-level retrieval: the stand-in keys of the non-retrieved blocks of the selected clusters.  Their gradient goes to dQ

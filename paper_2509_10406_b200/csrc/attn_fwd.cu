@@ -665,6 +665,40 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
   return MUSE_OK;
 }
 
+// The far field alone, with the selection given (the backward of the dipole correction needs each query's far
+// log-sum-exp again, which the forward does not hand over): lse_far [B*Hq*N], o_far [B*Hq*N*D] fp32, sel_tmp
+// [B*Hq*N*m] scratch that receives a copy of the selection.
+template <class T, int D>
+static int far_fwd_again_t(const Dims& d, int dtype, const T* Q, const float* qbar, const int32_t* off_q, const int32_t* perm_q,
+                           const SummPtrs& sp, const int32_t* sel_in, int32_t* sel_tmp, float* o_far, float* lse_far, int* status,
+                           cudaStream_t st) {
+  const int pq = d.B * d.Hq;
+  prof_mark("k_far_defaults", st);
+  k_far_defaults<<<dim3(cdiv(d.N, 256), pq), 256, 0, st>>>(d, lse_far, sel_tmp);
+  MUSE_LAUNCH_OK();
+  if (d.SB == 0) return MUSE_OK;
+  if (far_fwd_tc_supported(d, dtype) && !path_forced(kForceFarSimt))
+    return far_fwd_tc(d, sp, Q, off_q, perm_q, sel_in, sel_tmp, o_far, lse_far, status, st);
+  const size_t fs = far_smem(d.Ck, D);
+  MUSE_CUDA_OK(cudaFuncSetAttribute(k_far_fwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)fs));
+  prof_mark("k_far_fwd", st);
+  k_far_fwd<T, D><<<dim3(d.Cq, d.SB, pq), kFarThreads, fs, st>>>(d, Q, qbar, off_q, perm_q, sp, sel_in, sel_tmp, o_far, lse_far);
+  MUSE_LAUNCH_OK();
+  return MUSE_OK;
+}
+
+int far_fwd_again(const Dims& d, int dtype, const void* Q, const float* qbar, const int32_t* off_q, const int32_t* perm_q,
+                  const SummPtrs& sp, const int32_t* sel_in, int32_t* sel_tmp, float* o_far, float* lse_far, int* status,
+                  cudaStream_t st) {
+  typedef __nv_bfloat16 bf;
+  if (dtype == MUSE_F32) {
+    if (d.D == 64) return far_fwd_again_t<float, 64>(d, dtype, (const float*)Q, qbar, off_q, perm_q, sp, sel_in, sel_tmp, o_far, lse_far, status, st);
+    return far_fwd_again_t<float, 128>(d, dtype, (const float*)Q, qbar, off_q, perm_q, sp, sel_in, sel_tmp, o_far, lse_far, status, st);
+  }
+  if (d.D == 64) return far_fwd_again_t<bf, 64>(d, dtype, (const bf*)Q, qbar, off_q, perm_q, sp, sel_in, sel_tmp, o_far, lse_far, status, st);
+  return far_fwd_again_t<bf, 128>(d, dtype, (const bf*)Q, qbar, off_q, perm_q, sp, sel_in, sel_tmp, o_far, lse_far, status, st);
+}
+
 int attn_fwd(const Dims& d, int dtype, const void* Q, const void* K, const void* V, const int32_t* assign_q,
              const float* qbar, const int32_t* off_k, const int32_t* perm_k, const void* summaries,
              const int32_t* sel_in, const int32_t* bsel_in, void* O, float* LSE, int32_t* sel_out, int32_t* bsel_out, void* ws,

@@ -90,3 +90,53 @@ def test_dipole_argument_rules():
     s0, s1 = mb.muse_workspace_bytes(p0), mb.muse_workspace_bytes(p1)
     assert s1[4] >= s0[4] + 7 * (w.Cq + w.Ck) * w.D * w.D * 4
     assert mb.muse_summaries_layout(p0)[7] == s0[4]
+
+
+# ------------------------------------------------------------------ backward through the dipole correction
+
+BWD_CASES = {
+    "tiny_f32": (CASES["tiny"].with_(m=0), True, True),
+    "tiny_f32_m2": (CASES["tiny"].with_(m=2), True, True),
+    "tiny_f32_m2_noncausal": (CASES["tiny"].with_(m=2), False, True),
+    "tiny_f32_m2_frozen": (CASES["tiny"].with_(m=2), True, False),
+    "gqa_bf16_d64": (CASES["gqa_bf16"].with_(B=1, Hq=4, Hkv=2, m=0), True, True),
+    "gqa_bf16_d64_m6": (CASES["gqa_bf16"].with_(B=1, Hq=4, Hkv=2, m=6), True, True),
+    "d128_bf16_m8": (CASES["d128"].with_(m=8), True, True),                             # tensor-core far field and key-side pass
+    "d128_f32_odd_ck_m5": (CASES["d128"].with_(dtype="f32", m=5, Hq=1, Hkv=1, N=1000, Cq=8, Ck=24, S=4), True, True),
+}
+
+
+@pytest.mark.parametrize("name", list(BWD_CASES))
+def test_dipole_backward_matches_oracle(name):
+    from paper_2509_10406_b200 import binding as mb
+    w, causal, agg = BWD_CASES[name]
+    gain = 128.0
+    c = Case(w, gain=gain)
+    qbar32 = c.qbar.astype(np.float32)
+    p = c.params(dipole=1, causal=causal, agg_grad=agg)
+    buf = mb.MuseBuffers(p, backward=True)
+    Q, K, V, dO = c.dev()
+    aq, qb = to_dev(c.a_q, "i"), to_dev(qbar32, "f32")
+    mb.muse_summarize(p, K, V, to_dev(c.a_k, "i"), qb, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
+    mb.muse_attn_fwd(p, Q, K, V, aq, qb, buf.off_k, buf.perm_k, buf.summaries, None, buf.O, buf.LSE, buf.sel, buf.ws)
+    assert mb.muse_status(buf.ws) == 0
+    mb.muse_attn_bwd(p, Q, K, V, buf.O, buf.LSE, dO, aq, qb, buf.off_k, buf.perm_k, buf.summaries, buf.sel, buf.dQ, buf.dK, buf.dV, buf.ws)
+    torch.cuda.synchronize()
+    assert mb.muse_status(buf.ws) == 0
+    sel = to_np(buf.sel)[..., :w.m]
+    dQ, dK, dV = to_np(buf.dQ), to_np(buf.dK), to_np(buf.dV)
+    kw = dict(sigma=c.sigma, S=w.S, Ck=w.Ck, m=w.m, causal=causal, sel=sel, agg_grad=agg)
+    args = (c.Q.astype(np.float64), c.K.astype(np.float64), c.V.astype(np.float64), c.dO.astype(np.float64), c.a_q, c.a_k,
+            qbar32.astype(np.float64))
+    eQ, eK, eV = orc.layer_backward(*args, dipole=1, **kw)
+    pQ, pK, pV = orc.layer_backward(*args, **kw)                 # without the correction
+    errs = dict(dQ=rel_err(dQ, eQ), dK=rel_err(dK, eK), dV=rel_err(dV, eV))
+    moved = dict(dQ=rel_err(pQ, eQ), dK=rel_err(pK, eK), dV=rel_err(pV, eV))
+    print(name, errs, "correction moves the gradients by", moved)
+    t = tol(w.dtype)
+    assert all(v <= t for v in errs.values()), errs
+    # the comparison must be able to see the dipole terms: where they exceed the tolerance, the GPU is on the right side
+    for key, got, e, plain in (("dQ", dQ, eQ, pQ), ("dK", dK, eK, pK), ("dV", dV, eV, pV)):
+        if moved[key] > 4 * t:
+            assert rel_err(got, e) < rel_err(got, plain), key
+    assert max(moved.values()) > 4 * t or w.dtype != "f32"
