@@ -99,9 +99,12 @@ typedef struct muse_params {
   uint64_t seed;                /* used by MUSE_INIT_STRIDED and MUSE_INIT_KMEANSPP                */
   int32_t sel_mode;             /* MUSE_SEL_*: rank clusters by the Eq. 6 score per query, or by
                                    the accumulated log-mass per (query cluster, block)            */
-  int32_t dipole;               /* 0 off; 1: untilted, pre-merged dipole correction of the far field
-                                   (Appendix "Error Analysis", "Dipole Correction"); forward only,
-                                   requires m == 0 as in the paper                                   */
+  int32_t dipole;               /* 0 off; 1: untilted dipole correction of the far field (Appendix
+                                   "Error Analysis", "Dipole Correction"): pre-merged with m == 0 as in
+                                   the paper; with m > 0 each query's correction is the merge over the
+                                   clusters it did not retrieve ("Compatibility with Retrieval"); 2: the
+                                   same with the shared covariance tilted at one point per query head
+                                   (muse_dipole_tilt_point).  Forward and backward; not with k2 > 0     */
   int32_t agg_grad;             /* 1: differentiate the tilted aggregation weights; 0: constants   */
   const int32_t* head_map;      /* HOST [Hq] -> kv head, or NULL for h * Hkv / Hq                  */
 } muse_params_t;
@@ -125,9 +128,10 @@ MUSE_API int muse_workspace_bytes(const muse_params_t* p, size_t out[6]);
  *                           fp32 mode: unused (same offset as off[4])
  *   off[4] nu        [e][D] fp32 (fp32 mode) or bf16 (bf16 mode)
  *   off[5], off[6]          K and V bucketed by (cluster, block), [B,Hkv,N,D] dtype
- *   off[7] cbar             dipole == 1 only: merged dipole matrices Cbar = sum_j p(j) Cov_0j(v,k),
- *                           [B,Hq,SB,Cq][D value dims][D key dims], fp32 (fp32 mode) or bf16; with
- *                           dipole == 0 nothing is stored there
+ *   off[7] cbar             dipole != 0 only: merged dipole matrices Cbar = sum_j p(j) Cov_j(v,k),
+ *                           [B,Hq,SB,Cq][D value dims][D key dims], fp32 (fp32 mode, or m > 0) or bf16,
+ *                           followed by the shared covariances, the centroid weights, their sums and the
+ *                           tilt points (muse_dipole_layout); with dipole == 0 nothing is stored there
  *   off[8] per-block set    k2 > 0 only: a second mu | beta | kappa | kappa_lo | nu group of the same shapes
  *                           and spacing as off[0..4], holding the summaries of each block alone (plane s =
  *                           the keys of block s), which the spatial block selection scores; with k2 == 0
@@ -230,6 +234,23 @@ MUSE_API int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K,
                   const int32_t* off_k, const int32_t* perm_k, const void* summaries,
                   const int32_t* sel, const int32_t* bsel, void* dQ, void* dK, void* dV,
                   void* ws, size_t ws_bytes, cudaStream_t stream);
+
+/* Dipole correction, optional parts (Appendix "Error Analysis").
+ * muse_dipole_tilt_point - dipole == 2 only ("Untilted (Partially Specialized) Covariances": the shared
+ *   covariance tilted at ONE point per query head instead of at zero): writes that point, the mean of the
+ *   head's query centroids weighted by the number of queries each holds (assign_q [B,Hq,N], qbar
+ *   [B,Hq,Cq,D], DEVICE), into the summaries buffer at muse_dipole_layout off[4] ([B,Hq,D] fp32).  It is an
+ *   INPUT of muse_summarize, which builds the covariances with the weights exp(sigma qstar . k) normalised
+ *   inside each (cluster, plane) set; a caller may store any other tilt point there instead.  Call it (or
+ *   fill the array) before muse_summarize; muse_attn_bwd with summaries == NULL calls it itself.
+ * muse_dipole_layout - byte offsets inside the summaries buffer of: off[0] merged matrices Cbar
+ *   [B,Hq,SB,Cq][D][D] (fp32 when m > 0 or in fp32 mode, else bf16), off[1] shared covariances Cov
+ *   [B,H,SB,Ck][D value dims][D key dims] (H = Hkv for dipole == 1, Hq for dipole == 2; dtype), off[2]
+ *   centroid weights p [B,Hq,SB,Cq,Ck] (dtype), off[3] the sums over j of the stored weights [B,Hq,SB,Cq]
+ *   fp32, off[4] tilt points [B,Hq,D] fp32.  All outputs of muse_summarize except off[4]. */
+MUSE_API int muse_dipole_layout(const muse_params_t* p, size_t off[5]);
+MUSE_API int muse_dipole_tilt_point(const muse_params_t* p, const int32_t* assign_q, const float* qbar,
+                                    void* summaries, cudaStream_t stream);
 
 /* Seeded k-means++ start points, drawn on the GPU (the paper starts from a strided sample, Appendix
  * "Centroid Computation" step 1; this is the usual better-spread alternative for the Lloyd iterations).

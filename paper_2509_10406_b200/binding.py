@@ -23,7 +23,7 @@ MUSE_INIT_INDICES, MUSE_INIT_STRIDED, MUSE_INIT_CENTRES, MUSE_INIT_KMEANSPP = 0,
 
 EXPORTS = ("muse_workspace_bytes", "muse_summaries_layout", "muse_cluster", "muse_summarize",
            "muse_attn_fwd", "muse_attn_bwd", "muse_stream_workspace_bytes", "muse_stream_kmeans", "muse_balanced_assign",
-           "muse_kmeanspp_init",
+           "muse_kmeanspp_init", "muse_dipole_layout", "muse_dipole_tilt_point",
            "muse_cluster_streaming", "muse_cluster_noalloc", "muse_cluster_noalloc_max_bytes",
            "muse_cluster_noalloc_status_copy", "muse_status_copy", "muse_test_force_paths",
            "muse_test_wait_timeout", "muse_debug_report", "muse_profile", "muse_profile_report", "muse_strerror")
@@ -210,6 +210,18 @@ def muse_stream_kmeans(p, X, side, totals, counts, centres, ws, beta=0.9, first_
                                     ws.numel() * ws.element_size(), _stream()), "muse_stream_kmeans")
 
 
+def muse_dipole_layout(p):
+    """Byte offsets (cbar, cov, pw, zall, qstar) of the dipole arrays inside the summaries buffer."""
+    off = (ctypes.c_size_t * 5)()
+    _check(lib().muse_dipole_layout(ctypes.byref(p), off), "muse_dipole_layout")
+    return [int(x) for x in off]
+
+
+def muse_dipole_tilt_point(p, assign_q, qbar, summaries):
+    _check(lib().muse_dipole_tilt_point(ctypes.byref(p), _ptr(assign_q), _ptr(qbar), _ptr(summaries), _stream()),
+           "muse_dipole_tilt_point")
+
+
 def muse_kmeanspp_init(p, X, side, idx_out, ws):
     _check(lib().muse_kmeanspp_init(ctypes.byref(p), _ptr(X), int(side), _ptr(idx_out), _ptr(ws),
                                     ws.numel() * ws.element_size(), _stream()), "muse_kmeanspp_init")
@@ -308,6 +320,8 @@ class MuseBuffers:
 def muse_layer_forward(p, buf: MuseBuffers, Q, K, V, init_q=None, init_k=None, sel_in=None):
     """cluster -> summarize -> attention forward on the current stream."""
     muse_cluster(p, Q, K, init_q, init_k, buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, buf.ws)
+    if p.dipole == 2:
+        muse_dipole_tilt_point(p, buf.assign_q, buf.qbar, buf.summaries)
     muse_summarize(p, K, V, buf.assign_k, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
     muse_attn_fwd(p, Q, K, V, buf.assign_q, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, sel_in, buf.O, buf.LSE,
                   buf.sel, buf.ws, bsel_out=buf.bsel)

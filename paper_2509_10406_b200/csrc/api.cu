@@ -38,7 +38,7 @@ int resolve(const muse_params_t* p, Dims* d) {
   if (p->n_blocks < 0 || p->k2 < 0) return MUSE_ERR_INVALID_ARG;
   if (p->D != 64 && p->D != 128) return MUSE_ERR_UNSUPPORTED;
   if (p->Hq > kMaxHeads || p->m > kMaxM || p->Cq > kMaxC || p->Ck > kMaxC) return MUSE_ERR_UNSUPPORTED;
-  if (p->dipole != 0 && p->dipole != 1) return MUSE_ERR_INVALID_ARG;
+  if (p->dipole < 0 || p->dipole > 2) return MUSE_ERR_INVALID_ARG;
   if (p->k2 > 8 || (p->k2 > 0 && p->dipole != 0)) return MUSE_ERR_UNSUPPORTED;
   int S = p->causal ? (p->n_blocks == 0 ? 8 : p->n_blocks) : 1;
   if (p->N % S != 0) return MUSE_ERR_INVALID_ARG;
@@ -157,6 +157,28 @@ int muse_summaries_layout(const muse_params_t* p, size_t off[9]) {
   SummLayout L = summ_layout(d, p->dtype);
   off[0] = L.mu; off[1] = L.beta; off[2] = L.khi; off[3] = L.klo; off[4] = L.nu; off[5] = L.Kp; off[6] = L.Vp; off[7] = L.cbar; off[8] = L.blk;
   return MUSE_OK;
+}
+
+int muse_dipole_layout(const muse_params_t* p, size_t off[5]) {
+  Dims d;
+  int rc = resolve(p, &d);
+  if (rc != MUSE_OK) return rc;
+  if (off == nullptr) return MUSE_ERR_INVALID_ARG;
+  SummLayout L = summ_layout(d, p->dtype);
+  off[0] = L.cbar; off[1] = L.cov; off[2] = L.pw; off[3] = L.zall; off[4] = L.qstar;
+  return MUSE_OK;
+}
+
+int muse_dipole_tilt_point(const muse_params_t* p, const int32_t* assign_q, const float* qbar, void* summaries,
+                           cudaStream_t stream) {
+  Dims d;
+  int rc = resolve(p, &d);
+  if (rc != MUSE_OK) return rc;
+  if (!assign_q || !qbar || !summaries || !aligned16(qbar) || !aligned16(summaries)) return MUSE_ERR_INVALID_ARG;
+  if (d.dipole != 2) return MUSE_ERR_INVALID_ARG;
+  rc = dipole_tilt_point(d, assign_q, qbar, dipole_ptrs(summ_layout(d, p->dtype), summaries).qstar, stream);
+  prof_mark(nullptr, stream);
+  return rc;
 }
 
 int muse_cluster(const muse_params_t* p, const void* Q, const void* K, const int32_t* init_q,
@@ -343,6 +365,10 @@ int muse_attn_bwd(const muse_params_t* p, const void* Q, const void* K, const vo
     // Rebuild the summaries from the bucketed keys in the tail of the workspace (the keys keep the
     // bucketing that off_k / perm_k describe, so no sort is needed).
     char* tail = (char*)ws + need[3];
+    if (d.dipole == 2) {                                  // the rebuilt buffer needs its tilt point first
+      rc = dipole_tilt_point(d, assign_q, qbar, dipole_ptrs(summ_layout(d, p->dtype), tail).qstar, stream);
+      if (rc != MUSE_OK) return rc;
+    }
     rc = summarize(d, p->dtype, K, V, nullptr, qbar, const_cast<int32_t*>(off_k), const_cast<int32_t*>(perm_k), nullptr, nullptr,
                    nullptr, tail, tail + need[4], (int32_t*)ws, stream);
     if (rc != MUSE_OK) return rc;

@@ -820,7 +820,7 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
     }
     MUSE_LAUNCH_OK();
     if (d.dipole) {
-      rc = dipole_bwd_keys(d, dtype, Kp, Vp, off_k, w.dip, w.dK_perm, w.dV_perm, st);
+      rc = dipole_bwd_keys(d, dtype, Kp, Vp, off_k, dipole_ptrs(L, base), w.dip, w.dK_perm, w.dV_perm, st);
       if (rc != MUSE_OK) return rc;
     }
   }

@@ -22,7 +22,8 @@ struct Dims {
   int SB;       // stored summary planes: S-1 (causal) or 1
   int Bs;       // block size N / S
   int causal, sel_mode, agg_grad;
-  int dipole;   // 1: untilted dipole correction of the far field; with m > 0 restricted to the clusters a query did not retrieve
+  int dipole;   // 1: untilted dipole correction of the far field; with m > 0 restricted to the clusters a query did not retrieve;
+                // 2: the same with the shared covariance tilted at one point per query head (kept in the summaries buffer)
   int k2;       // spatial selection: 0 = every earlier block of a selected cluster is retrieved; > 0 = only the k2 best (causal only)
   float sigma;
   HeadMap hm;
@@ -184,7 +185,7 @@ int split_qbar(const Dims& d, const float* qbar, void* qhi, void* qlo, cudaStrea
 //   cbar (dipole only): merged dipole matrices [B,Hq,SB,Cq][D value dims][D key dims], fp32 or bf16
 //   blk (k2 > 0 only): a second set mu | beta | kappa (hi, lo) | nu with the same shapes holding the PER-BLOCK
 //              (pre-accumulation) summaries: plane s = the summary of the keys of block s alone
-struct SummLayout { size_t mu, beta, khi, klo, nu, Kp, Vp, cbar, cov, pw, zall, blk, blk_beta, blk_khi, blk_klo, blk_nu, total; };
+struct SummLayout { size_t mu, beta, khi, klo, nu, Kp, Vp, cbar, cov, pw, zall, qstar, blk, blk_beta, blk_khi, blk_klo, blk_nu, total; };
 SummLayout summ_layout(const Dims& d, int dtype);
 
 struct SummPtrs { float* mu; float* beta; void* khi; void* klo; void* nu; };
@@ -193,10 +194,10 @@ inline SummPtrs summ_ptrs(const SummLayout& L, const void* base_) {
   return SummPtrs{(float*)(b + L.mu), (float*)(b + L.beta), b + L.khi, b + L.klo, b + L.nu};
 }
 // dipole part of the summaries buffer: merged matrices, shared covariances, centroid weights and their sums
-struct DipolePtrs { void* cbar; void* cov; void* pw; float* zall; };
+struct DipolePtrs { void* cbar; void* cov; void* pw; float* zall; float* qstar; };
 inline DipolePtrs dipole_ptrs(const SummLayout& L, const void* base_) {
   char* b = (char*)base_;
-  return DipolePtrs{b + L.cbar, b + L.cov, b + L.pw, (float*)(b + L.zall)};
+  return DipolePtrs{b + L.cbar, b + L.cov, b + L.pw, (float*)(b + L.zall), (float*)(b + L.qstar)};
 }
 inline SummPtrs summ_ptrs_blk(const SummLayout& L, const void* base_) {      // the per-block set (k2 > 0)
   char* b = (char*)base_;
@@ -208,6 +209,7 @@ size_t dipole_fwd_ws_bytes(const Dims& d);
 struct DipoleBwdWs { int32_t* sel_tmp; float *lse_far, *zq, *dz, *delta_far, *xq, *corr, *csub, *dcbar, *dcov, *dpw, *dzs; };
 DipoleBwdWs dipole_bwd_ws(const Dims& d, Arena& ar);
 bool dipole_bwd_supported(const Dims& d);
+int dipole_tilt_point(const Dims& d, const int32_t* assign_q, const float* qbar, float* qstar, cudaStream_t st);
 int far_fwd_again(const Dims& d, int dtype, const void* Q, const float* qbar, const int32_t* off_q, const int32_t* perm_q,
                   const SummPtrs& sp, const int32_t* sel_in, int32_t* sel_tmp, float* o_far, float* lse_far, int* status,
                   cudaStream_t st);
@@ -216,8 +218,8 @@ int dipole_bwd_pre(const Dims& d, int dtype, const void* Q, const void* dO, cons
                    const int32_t* pairs, const DipoleBwdWs& w, float* dQacc, cudaStream_t st);
 int dipole_bwd_dmu(const Dims& d, int dtype, const DipolePtrs& dp, const DipoleBwdWs& w, float* dS, int grad_by_key_cluster,
                    cudaStream_t st);
-int dipole_bwd_keys(const Dims& d, int dtype, const void* Kp, const void* Vp, const int32_t* off_k, const DipoleBwdWs& w,
-                    float* dK_perm, float* dV_perm, cudaStream_t st);
+int dipole_bwd_keys(const Dims& d, int dtype, const void* Kp, const void* Vp, const int32_t* off_k, const DipolePtrs& dp,
+                    const DipoleBwdWs& w, float* dK_perm, float* dV_perm, cudaStream_t st);
 int dipole_build(const Dims& d, int dtype, const void* Kp, const void* Vp, const int32_t* off_k, const float* mu,
                  const DipolePtrs& dp, int* status, cudaStream_t st);
 int dipole_apply(const Dims& d, int dtype, const void* Q, const float* qbar, const int32_t* assign_q, const int32_t* off_q,

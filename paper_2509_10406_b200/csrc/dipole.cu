@@ -29,19 +29,27 @@ int dipole_merge_tc(const Dims& d, const void* P, const void* cov, void* cbar, i
 // moments small.  Thread (ty, tx) owns a TV x TV sub-block: value dims ty*TV.., key dims tx*TV...
 constexpr int kCovKeys = 8;
 
-template <class T, class ST, int D>
+// TILT (dipole == 2): one covariance set per QUERY head, its members weighted by w_u ~ exp(sigma qstar . k_u) with
+// qstar the head's shared tilt point; the weights are carried relative to a running maximum of the logits and all
+// running moments are rescaled when it grows.
+template <class T, class ST, int D, bool TILT>
 __global__ void __launch_bounds__(256)
 k_dipole_cov(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const int32_t* __restrict__ off_k,
-             ST* __restrict__ cov) {
+             const float* __restrict__ qstar, ST* __restrict__ cov) {
   constexpr int TV = D / 16;
-  __shared__ float ks[kCovKeys][D], vs[kCovKeys][D], k0[D];
-  const int j = blockIdx.x, pk = blockIdx.y, tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  __shared__ float ks[kCovKeys][D], vs[kCovKeys][D], k0[D], qs_[D], wl[kCovKeys];
+  const int j = blockIdx.x, pc = blockIdx.y, tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const int pk = TILT ? (pc / dm.Hq) * dm.Hkv + dm.hm.g[pc % dm.Hq] : pc;
   const int32_t* off = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const T* Kb = Kp + (size_t)pk * dm.N * D;
   const T* Vb = Vp + (size_t)pk * dm.N * D;
   const int first = off[0];
-  if (tid < D) k0[tid] = first < off[dm.S] ? to_f(Kb[(size_t)first * D + tid]) : 0.f;
+  if (tid < D) {
+    k0[tid] = first < off[dm.S] ? to_f(Kb[(size_t)first * D + tid]) : 0.f;
+    qs_[tid] = TILT ? dm.sigma * qstar[(size_t)pc * D + tid] : 0.f;
+  }
   float A[TV][TV], sv[TV], sk[TV];
+  float wsum = 0.f, wmax = -INFINITY;             // TILT: sum of the weights, and the logit they are relative to
 #pragma unroll
   for (int a = 0; a < TV; ++a) {
     sv[a] = 0.f; sk[a] = 0.f;
@@ -64,22 +72,47 @@ k_dipole_cov(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const 
         }
       }
       __syncthreads();
+      if (TILT) {
+        // logits of the chunk's keys (shifted keys: a constant per cluster, which cancels in the normalised weights)
+        const int wq = tid >> 5, ln = tid & 31;
+        float l = 0.f;
+        if (wq < nk)
+          for (int c = ln; c < D; c += 32) l = fmaf(qs_[c], ks[wq][c], l);
+        l = warp_sum(l);
+        if (ln == 0) wl[wq] = wq < nk ? l : -INFINITY;
+        __syncthreads();
+        float mx = wmax;
+        for (int r = 0; r < nk; ++r) mx = fmaxf(mx, wl[r]);
+        if (mx > wmax) {
+          const float f = wmax == -INFINITY ? 0.f : expf(wmax - mx);
+          wsum *= f;
+#pragma unroll
+          for (int a = 0; a < TV; ++a) {
+            sv[a] *= f; sk[a] *= f;
+#pragma unroll
+            for (int c = 0; c < TV; ++c) A[a][c] *= f;
+          }
+          wmax = mx;
+        }
+      }
       for (int r = 0; r < nk; ++r) {
+        const float wr = TILT ? expf(wl[r] - wmax) : 1.f;
         float kv_[TV], vv_[TV];
 #pragma unroll
-        for (int a = 0; a < TV; ++a) { kv_[a] = ks[r][tx * TV + a]; vv_[a] = vs[r][ty * TV + a]; }
+        for (int a = 0; a < TV; ++a) { kv_[a] = ks[r][tx * TV + a]; vv_[a] = wr * vs[r][ty * TV + a]; }
 #pragma unroll
         for (int a = 0; a < TV; ++a) {
-          sv[a] += vv_[a]; sk[a] += kv_[a];
+          sv[a] += vv_[a]; sk[a] = fmaf(wr, kv_[a], sk[a]);
 #pragma unroll
           for (int c = 0; c < TV; ++c) A[a][c] = fmaf(vv_[a], kv_[c], A[a][c]);
         }
+        wsum += wr;
       }
       n += nk;
     }
     // centred covariance of everything seen so far = what queries of block pl + 1 see
-    const float inv = n > 0 ? 1.f / (float)n : 0.f;
-    ST* out = cov + (((size_t)pk * dm.SB + pl) * dm.Ck + j) * D * D;
+    const float inv = n > 0 ? 1.f / (TILT ? wsum : (float)n) : 0.f;
+    ST* out = cov + (((size_t)pc * dm.SB + pl) * dm.Ck + j) * D * D;
 #pragma unroll
     for (int a = 0; a < TV; ++a) {
       const float vm = sv[a] * inv;
@@ -128,7 +161,7 @@ k_dipole_merge(Dims dm, const ST* __restrict__ P, const ST* __restrict__ cov, OT
   const int DD = dm.D * dm.D;
   const int x = blockIdx.x * 256 + threadIdx.x, i0 = blockIdx.y * kMrgI;
   const int pp = blockIdx.z, pq = pp / dm.SB, pl = pp % dm.SB;
-  const int pk = (pq / dm.Hq) * dm.Hkv + dm.hm.g[pq % dm.Hq];
+  const int pk = dm.dipole == 2 ? pq : (pq / dm.Hq) * dm.Hkv + dm.hm.g[pq % dm.Hq];     // head that owns the covariances
   const ST* Pb = P + ((size_t)pp * dm.Cq) * dm.Ck;
   const ST* cb = cov + (((size_t)pk * dm.SB + pl) * dm.Ck) * DD;
   float acc[kMrgI];
@@ -293,6 +326,35 @@ k_dipole_apply(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar,
   }
 }
 
+// ---- the shared tilt point of dipole == 2: the mean of a head's query centroids weighted by their member counts ----
+// ("Untilted (Partially Specialized) Covariances": centring the shared tilt at the mass-weighted mean query centroid.)
+// One CTA per query head: integer histogram of the assignments, then a fixed-order weighted sum.
+__global__ void __launch_bounds__(256)
+k_dipole_qstar(Dims dm, const int32_t* __restrict__ assign_q, const float* __restrict__ qbar, float* __restrict__ qstar) {
+  __shared__ int cnt[kMaxC];
+  const int pq = blockIdx.x, tid = threadIdx.x;
+  for (int i = tid; i < dm.Cq; i += 256) cnt[i] = 0;
+  __syncthreads();
+  const int32_t* aq = assign_q + (size_t)pq * dm.N;
+  for (int t = tid; t < dm.N; t += 256) {
+    const int i = aq[t];
+    if (MUSE_IN_RANGE(i, dm.Cq)) atomicAdd(&cnt[i], 1);
+  }
+  __syncthreads();
+  for (int c = tid; c < dm.D; c += 256) {
+    float s = 0.f;
+    for (int i = 0; i < dm.Cq; ++i) s = fmaf((float)cnt[i], qbar[((size_t)pq * dm.Cq + i) * dm.D + c], s);
+    qstar[(size_t)pq * dm.D + c] = s / (float)dm.N;
+  }
+}
+
+int dipole_tilt_point(const Dims& d, const int32_t* assign_q, const float* qbar, float* qstar, cudaStream_t st) {
+  prof_mark("k_dipole_qstar", st);
+  k_dipole_qstar<<<d.B * d.Hq, 256, 0, st>>>(d, assign_q, qbar, qstar);
+  MUSE_LAUNCH_OK();
+  return MUSE_OK;
+}
+
 // ---- host side ------------------------------------------------------------------------------------
 // Scratch of the forward pass (and of the backward's recomputation): the retrieved clusters' rows.
 size_t dipole_fwd_ws_bytes(const Dims& d) {
@@ -307,7 +369,8 @@ static int dipole_build_t(const Dims& d, int dtype, const T* Kp, const T* Vp, co
                           const DipolePtrs& dp, int* status, cudaStream_t st) {
   ST* cov = (ST*)dp.cov; ST* P = (ST*)dp.pw;
   prof_mark("k_dipole_cov", st);
-  k_dipole_cov<T, ST, D><<<dim3(d.Ck, d.B * d.Hkv), 256, 0, st>>>(d, Kp, Vp, off_k, cov);
+  if (d.dipole == 2) k_dipole_cov<T, ST, D, true><<<dim3(d.Ck, d.B * d.Hq), 256, 0, st>>>(d, Kp, Vp, off_k, dp.qstar, cov);
+  else k_dipole_cov<T, ST, D, false><<<dim3(d.Ck, d.B * d.Hkv), 256, 0, st>>>(d, Kp, Vp, off_k, nullptr, cov);
   MUSE_LAUNCH_OK();
   const long long rows = (long long)d.B * d.Hq * d.SB * d.Cq;
   prof_mark("k_dipole_weights", st);

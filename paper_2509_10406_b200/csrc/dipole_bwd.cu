@@ -14,6 +14,9 @@
 //   log-masses     dmu_ijb  = p (dp - sum_k p_k dp_k)                  -> added to the summary gradient of the monopole
 //   keys, values   Cov_jb = mean((v - vm)(k - km)^T) over blocks <= b of cluster j:
 //                  dV_u = sum_{b >= block(u)} dCov_jb (k_u - km_b) / n_b,  dK_u = sum_b dCov_jb^T (v_u - vm_b) / n_b.
+//                  dipole == 2 (weights w_ub = exp(l_u - lse_b), l_u = sigma qstar.k_u, in place of 1 / n_b): the same
+//                  with w_ub, plus, unless agg_grad = 0, dl_u = sum_b w_ub [(v_u - vm_b)^T dCov_jb (k_u - km_b)
+//                  - <dCov_jb, Cov_jb>] and dK_u += sigma qstar dl_u.
 // Kernels: k_dipole_bwd_prep (per query), k_dipole_bwd_seg (per query segment), k_dipole_bwd_pairs (per group of the
 // retrieval's inverse index, m > 0), k_dipole_dcov / k_dipole_dpw (the two dense contractions over the query and key
 // clusters), k_dipole_dmu (softmax backward), k_dipole_cov_bwd (per key cluster: suffix sums over planes, then one
@@ -326,10 +329,16 @@ __global__ void k_dipole_dmu(Dims dm, const ST* __restrict__ P, const float* __r
 }
 
 // ---- through the covariances to keys and values: one CTA per (key cluster, query head) ----------------------------
-template <class T, int D>
+// With w_ub = f_u / W_b (f_u = exp(l_u - max logit of the cluster), W_b = sum of f over the plane's members):
+//   dV_u = f_u (A k_u - a_k),  dK_u = f_u (A^T v_u - a_v),  A = sum_{b >= block(u)} dCov_b / W_b,
+//   a_k = sum_b dCov_b km_b / W_b,  a_v = sum_b dCov_b^T vm_b / W_b,
+//   dl_u = f_u (v_u.(A k_u - a_k) - a_v.k_u + s),  s = sum_b (vm_b^T dCov_b km_b - <dCov_b, Cov_b>) / W_b
+// (untilted: f = 1, W_b = n_b, no dl).  Keys enter shifted by the cluster's first key, which changes none of these.
+template <class T, class ST, int D, bool TILT>
 __global__ void __launch_bounds__(256)
 k_dipole_cov_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, const int32_t* __restrict__ off_k,
-                 const float* __restrict__ dcov, float* __restrict__ dK_perm, float* __restrict__ dV_perm) {
+                 const float* __restrict__ dcov, const float* __restrict__ qstar, const ST* __restrict__ cov,
+                 float* __restrict__ dK_perm, float* __restrict__ dV_perm) {
   extern __shared__ float smd[];
   float* As = smd;                              // As[dv][dk], pitch D + 1: sum over later planes of dCov / n
   float* Gs = As + D * (D + 1);                 // this plane's dCov / n
@@ -340,32 +349,63 @@ k_dipole_cov_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, co
   float* ak = vs + kDbQ * D;                    // [D] sum of dCov km / n
   float* av = ak + D;                           // [D] sum of dCov^T vm / n
   float* k0 = av + D;
-  const int j = blockIdx.x, pq = blockIdx.y, tid = threadIdx.x;
+  float* qs_ = k0 + D;                          // [D] sigma * tilt point
+  float* wb = qs_ + D;                          // [SB] W_b
+  __shared__ float red[8], fk[kDbQ], dl_s[kDbQ], s_suf, lmax_s;
+  const int j = blockIdx.x, pq = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int pk = (pq / dm.Hq) * dm.Hkv + dm.hm.g[pq % dm.Hq];
   const int32_t* off = off_k + (size_t)pk * (dm.Ck * dm.S + 1) + (size_t)j * dm.S;
   const T* Kb = Kp + (size_t)pk * dm.N * D;
   const T* Vb = Vp + (size_t)pk * dm.N * D;
   const int first = off[0];
   if (first >= off[dm.SB]) return;              // no key of this cluster is visible to anyone
-  if (tid < D) { k0[tid] = to_f(Kb[(size_t)first * D + tid]); ak[tid] = 0.f; av[tid] = 0.f; }
+  if (tid < D) {
+    k0[tid] = to_f(Kb[(size_t)first * D + tid]); ak[tid] = 0.f; av[tid] = 0.f;
+    qs_[tid] = TILT ? dm.sigma * qstar[(size_t)pq * D + tid] : 0.f;
+  }
   for (int e = tid; e < D * (D + 1); e += 256) As[e] = 0.f;
+  if (tid == 0) { s_suf = 0.f; lmax_s = 0.f; }
   __syncthreads();
-  // prefix means per plane (plane pl = blocks 0..pl)
+  // logit of a key relative to the cluster's first key: one warp, all lanes return it
+  auto logit = [&](int u) {
+    float l = 0.f;
+    for (int c = lane; c < D; c += 32) l = fmaf(qs_[c], to_f(Kb[(size_t)u * D + c]) - k0[c], l);
+    return warp_sum(l);
+  };
+  if (TILT) {                                   // largest logit over the visible members
+    float mx = -INFINITY;
+    for (int u = first + warp; u < off[dm.SB]; u += 8) mx = fmaxf(mx, logit(u));
+    if (lane == 0) red[warp] = mx;
+    __syncthreads();
+    if (tid == 0) { float m = red[0]; for (int w = 1; w < 8; ++w) m = fmaxf(m, red[w]); lmax_s = m; }
+    __syncthreads();
+  }
+  const float lmax = lmax_s;
+  // prefix means per plane (plane pl = blocks 0..pl), weighted by f_u
   if (tid < 2 * D) {
     const bool isv = tid >= D;
     const int c = tid % D;
-    float s = 0.f;
+    float s = 0.f, wsum = 0.f;
     for (int pl = 0; pl < dm.SB; ++pl) {
-      for (int u = off[pl]; u < off[pl + 1]; ++u) s += isv ? to_f(Vb[(size_t)u * D + c]) : to_f(Kb[(size_t)u * D + c]) - k0[c];
-      const int n = off[pl + 1] - first;
-      (isv ? vb : kb)[pl * D + c] = n > 0 ? s / (float)n : 0.f;
+      for (int u = off[pl]; u < off[pl + 1]; ++u) {
+        float f = 1.f;
+        if (TILT) {                             // every thread recomputes the key's weight (a cluster has few keys)
+          float l = 0.f;
+          for (int cc = 0; cc < D; ++cc) l = fmaf(qs_[cc], to_f(Kb[(size_t)u * D + cc]) - k0[cc], l);
+          f = expf(l - lmax);
+        }
+        s = fmaf(f, isv ? to_f(Vb[(size_t)u * D + c]) : to_f(Kb[(size_t)u * D + c]) - k0[c], s);
+        wsum += f;
+      }
+      (isv ? vb : kb)[pl * D + c] = wsum > 0.f ? s / wsum : 0.f;
+      if (tid == 0) wb[pl] = wsum;
     }
   }
   __syncthreads();
   for (int pl = dm.SB - 1; pl >= 0; --pl) {
-    const int n = off[pl + 1] - first;
-    if (n > 0) {
-      const float inv = 1.f / (float)n;
+    const float n = wb[pl];
+    if (n > 0.f) {
+      const float inv = 1.f / n;
       const float* g = dcov + (((size_t)pq * dm.SB + pl) * dm.Ck + j) * D * D;
       for (int e = tid; e < D * D / 4; e += 256) {
         const int dv = e / (D / 4), c4 = (e % (D / 4)) * 4;
@@ -379,11 +419,22 @@ k_dipole_cov_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, co
         float s = 0.f;
         for (int dk = 0; dk < D; ++dk) s = fmaf(Gs[tid * (D + 1) + dk], kb[pl * D + dk], s);
         ak[tid] += s;
+        if (TILT && dm.agg_grad) {              // vm^T (dCov / W) km, over the D value dims
+          const float part = warp_sum(s * vb[pl * D + tid]);
+          if (lane == 0) atomicAdd(&s_suf, part);
+        }
       } else if (tid < 2 * D) {
         const int dk = tid - D;
         float s = 0.f;
         for (int dv = 0; dv < D; ++dv) s = fmaf(Gs[dv * (D + 1) + dk], vb[pl * D + dv], s);
         av[dk] += s;
+      }
+      if (TILT && dm.agg_grad) {                // - <dCov / W, Cov> with the stored covariance
+        const ST* cv = cov + (((size_t)pq * dm.SB + pl) * dm.Ck + j) * D * D;
+        float part = 0.f;
+        for (int e = tid; e < D * D; e += 256) part = fmaf(Gs[(e / D) * (D + 1) + e % D], to_f(cv[e]), part);
+        part = warp_sum(part);
+        if (lane == 0) atomicAdd(&s_suf, -part);
       }
     }
     __syncthreads();
@@ -395,8 +446,12 @@ k_dipole_cov_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, co
         ks[e] = r < nk ? to_f(Kb[(size_t)(u0 + r) * D + c]) - k0[c] : 0.f;
         vs[e] = r < nk ? to_f(Vb[(size_t)(u0 + r) * D + c]) : 0.f;
       }
+      if (warp < kDbQ) {
+        const float l = TILT && warp < nk ? logit(u0 + warp) : 0.f;
+        if (lane == 0) { fk[warp] = TILT ? (warp < nk ? expf(l - lmax) : 0.f) : 1.f; dl_s[warp] = 0.f; }
+      }
       __syncthreads();
-      if (tid < D) {                            // dV_u[dv] = sum_dk As[dv][dk] k_u[dk] - ak[dv]
+      if (tid < D) {                            // dV_u[dv] = f_u (sum_dk As[dv][dk] k_u[dk] - ak[dv])
         float acc[kDbQ];
 #pragma unroll
         for (int a = 0; a < kDbQ; ++a) acc[a] = -ak[tid];
@@ -405,8 +460,15 @@ k_dipole_cov_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, co
 #pragma unroll
           for (int a = 0; a < kDbQ; ++a) acc[a] = fmaf(c, ks[a * D + dk], acc[a]);
         }
-        for (int a = 0; a < nk; ++a) dV_perm[((size_t)pq * dm.N + u0 + a) * D + tid] += acc[a];
-      } else if (tid < 2 * D) {                 // dK_u[dk] = sum_dv As[dv][dk] v_u[dv] - av[dk]
+        for (int a = 0; a < nk; ++a) dV_perm[((size_t)pq * dm.N + u0 + a) * D + tid] += fk[a] * acc[a];
+        if (TILT && dm.agg_grad) {
+#pragma unroll
+          for (int a = 0; a < kDbQ; ++a) {      // v_u.(A k_u - a_k) - a_v.k_u  (D == value dims == key dims)
+            const float part = warp_sum(vs[a * D + tid] * acc[a] - av[tid] * ks[a * D + tid]);
+            if (lane == 0) atomicAdd(&dl_s[a], part);
+          }
+        }
+      } else if (tid < 2 * D) {                 // dK_u[dk] = f_u (sum_dv As[dv][dk] v_u[dv] - av[dk])
         const int dk = tid - D;
         float acc[kDbQ];
 #pragma unroll
@@ -416,7 +478,12 @@ k_dipole_cov_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, co
 #pragma unroll
           for (int a = 0; a < kDbQ; ++a) acc[a] = fmaf(c, vs[a * D + dv], acc[a]);
         }
-        for (int a = 0; a < nk; ++a) dK_perm[((size_t)pq * dm.N + u0 + a) * D + dk] += acc[a];
+        for (int a = 0; a < nk; ++a) dK_perm[((size_t)pq * dm.N + u0 + a) * D + dk] += fk[a] * acc[a];
+      }
+      __syncthreads();
+      if (TILT && dm.agg_grad && tid < D) {     // dK_u += sigma qstar dl_u
+        const float s = s_suf;
+        for (int a = 0; a < nk; ++a) dK_perm[((size_t)pq * dm.N + u0 + a) * D + tid] += qs_[tid] * fk[a] * (dl_s[a] + s);
       }
       __syncthreads();
     }
@@ -444,8 +511,8 @@ DipoleBwdWs dipole_bwd_ws(const Dims& d, Arena& ar) {
 }
 
 bool dipole_bwd_supported(const Dims& d) {
-  const size_t smem = (size_t)(2 * d.D * (d.D + 1) + 2 * d.SB * d.D + 2 * kDbQ * d.D + 3 * d.D) * sizeof(float);
-  return d.dipole == 1 && smem <= 200 * 1024;
+  const size_t smem = (size_t)(2 * d.D * (d.D + 1) + 2 * d.SB * d.D + 2 * kDbQ * d.D + 4 * d.D + d.SB) * sizeof(float);
+  return smem <= 200 * 1024;
 }
 
 // Before the far-field backward: corr, zq, lse_far are the forward's correction, weight sum and far log-sum-exp.
@@ -519,27 +586,33 @@ int dipole_bwd_dmu(const Dims& d, int dtype, const DipolePtrs& dp, const DipoleB
   return MUSE_OK;
 }
 
-template <class T, int D>
-static int dipole_bwd_keys_t(const Dims& d, const T* Kp, const T* Vp, const int32_t* off_k, const DipoleBwdWs& w, float* dK_perm,
-                             float* dV_perm, cudaStream_t st) {
-  const size_t smem = (size_t)(2 * D * (D + 1) + 2 * d.SB * D + 2 * kDbQ * D + 3 * D) * sizeof(float);
-  MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_cov_bwd<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+template <class T, class ST, int D>
+static int dipole_bwd_keys_t(const Dims& d, const T* Kp, const T* Vp, const int32_t* off_k, const DipolePtrs& dp, const DipoleBwdWs& w,
+                             float* dK_perm, float* dV_perm, cudaStream_t st) {
+  const size_t smem = (size_t)(2 * D * (D + 1) + 2 * d.SB * D + 2 * kDbQ * D + 4 * D + d.SB) * sizeof(float);
+  const dim3 grid(d.Ck, d.B * d.Hq);
   prof_mark("k_dipole_cov_bwd", st);
-  k_dipole_cov_bwd<T, D><<<dim3(d.Ck, d.B * d.Hq), 256, smem, st>>>(d, Kp, Vp, off_k, w.dcov, dK_perm, dV_perm);
+  if (d.dipole == 2) {
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_cov_bwd<T, ST, D, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k_dipole_cov_bwd<T, ST, D, true><<<grid, 256, smem, st>>>(d, Kp, Vp, off_k, w.dcov, dp.qstar, (const ST*)dp.cov, dK_perm, dV_perm);
+  } else {
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_cov_bwd<T, ST, D, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k_dipole_cov_bwd<T, ST, D, false><<<grid, 256, smem, st>>>(d, Kp, Vp, off_k, w.dcov, nullptr, (const ST*)dp.cov, dK_perm, dV_perm);
+  }
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }
 
 // After the key-side pass of the monopole: the covariances' gradient reaches the bucketed keys and values.
-int dipole_bwd_keys(const Dims& d, int dtype, const void* Kp, const void* Vp, const int32_t* off_k, const DipoleBwdWs& w,
-                    float* dK_perm, float* dV_perm, cudaStream_t st) {
+int dipole_bwd_keys(const Dims& d, int dtype, const void* Kp, const void* Vp, const int32_t* off_k, const DipolePtrs& dp,
+                    const DipoleBwdWs& w, float* dK_perm, float* dV_perm, cudaStream_t st) {
   typedef __nv_bfloat16 bf;
   if (dtype == MUSE_F32) {
-    if (d.D == 64) return dipole_bwd_keys_t<float, 64>(d, (const float*)Kp, (const float*)Vp, off_k, w, dK_perm, dV_perm, st);
-    return dipole_bwd_keys_t<float, 128>(d, (const float*)Kp, (const float*)Vp, off_k, w, dK_perm, dV_perm, st);
+    if (d.D == 64) return dipole_bwd_keys_t<float, float, 64>(d, (const float*)Kp, (const float*)Vp, off_k, dp, w, dK_perm, dV_perm, st);
+    return dipole_bwd_keys_t<float, float, 128>(d, (const float*)Kp, (const float*)Vp, off_k, dp, w, dK_perm, dV_perm, st);
   }
-  if (d.D == 64) return dipole_bwd_keys_t<bf, 64>(d, (const bf*)Kp, (const bf*)Vp, off_k, w, dK_perm, dV_perm, st);
-  return dipole_bwd_keys_t<bf, 128>(d, (const bf*)Kp, (const bf*)Vp, off_k, w, dK_perm, dV_perm, st);
+  if (d.D == 64) return dipole_bwd_keys_t<bf, bf, 64>(d, (const bf*)Kp, (const bf*)Vp, off_k, dp, w, dK_perm, dV_perm, st);
+  return dipole_bwd_keys_t<bf, bf, 128>(d, (const bf*)Kp, (const bf*)Vp, off_k, dp, w, dK_perm, dV_perm, st);
 }
 
 }  // namespace muse

@@ -35,7 +35,7 @@ k_dipole_merge_tc(Dims dm, const __grid_constant__ CUtensorMap tm_p, const __gri
   const int DD = dm.D * dm.D;
   const int x0 = blockIdx.x * kDmN, i0 = blockIdx.y * 256;
   const int pp = blockIdx.z, pq = pp / dm.SB, pl = pp % dm.SB;
-  const int pk = (pq / dm.Hq) * dm.Hkv + dm.hm.g[pq % dm.Hq];
+  const int pk = dm.dipole == 2 ? pq : (pq / dm.Hq) * dm.Hkv + dm.hm.g[pq % dm.Hq];   // head that owns the covariances
   const int halves = dm.Cq - i0 > 128 ? 2 : 1;
   const int rowA = pp * dm.Cq + i0;                              // first P row of this tile
   const int rowB = (pk * dm.SB + pl) * dm.Ck;                    // first covariance row of this (kv head, plane)
@@ -121,14 +121,14 @@ k_dipole_merge_tc(Dims dm, const __grid_constant__ CUtensorMap tm_p, const __gri
 
 bool dipole_merge_tc_supported(const Dims& d, int dtype) {
   // row coordinates of the tensor maps are 32-bit
-  const long long rows_p = (long long)d.B * d.Hq * d.SB * d.Cq, rows_c = (long long)d.B * d.Hkv * d.SB * d.Ck;
+  const long long rows_p = (long long)d.B * d.Hq * d.SB * d.Cq, rows_c = (long long)d.B * (d.dipole == 2 ? d.Hq : d.Hkv) * d.SB * d.Ck;
   return dtype == MUSE_BF16 && d.Ck % kDmK == 0 && (d.D * d.D) % kDmN == 0 && rows_p < (1ll << 31) && rows_c < (1ll << 31);
 }
 
 int dipole_merge_tc(const Dims& d, const void* P, const void* cov, void* cbar, int out_f32, int* status, cudaStream_t st) {
   CUtensorMap tp, tcv;
   int rc = make_tmap_bf16_rows(&tp, P, (uint64_t)d.B * d.Hq * d.SB * d.Cq, d.Ck, 128);
-  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tcv, cov, (uint64_t)d.B * d.Hkv * d.SB * d.Ck, d.D * d.D, kDmK);
+  if (rc == MUSE_OK) rc = make_tmap_bf16_rows(&tcv, cov, (uint64_t)d.B * (d.dipole == 2 ? d.Hq : d.Hkv) * d.SB * d.Ck, d.D * d.D, kDmK);
   if (rc != MUSE_OK) return rc;
   const size_t smem = (size_t)kDmStages * kDmStage + 1024;
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_merge_tc<bf16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

@@ -29,7 +29,8 @@ SummLayout summ_layout(const Dims& d, int dtype) {
   L.cov = up(L.cbar + (d.dipole ? (size_t)d.B * d.Hq * d.SB * d.Cq * d.D * d.D * ecb : 0));
   L.pw = up(L.cov + (d.dipole ? (size_t)d.B * covh * d.SB * d.Ck * d.D * d.D * es : 0));
   L.zall = up(L.pw + (d.dipole ? ent * es : 0));
-  L.blk = up(L.zall + (d.dipole ? (size_t)d.B * d.Hq * d.SB * d.Cq * sizeof(float) : 0));
+  L.qstar = up(L.zall + (d.dipole ? (size_t)d.B * d.Hq * d.SB * d.Cq * sizeof(float) : 0));
+  L.blk = up(L.qstar + (d.dipole == 2 ? (size_t)d.B * d.Hq * d.D * sizeof(float) : 0));
   L.blk_beta = L.blk_khi = L.blk_klo = L.blk_nu = L.blk;
   L.total = L.blk;
   if (d.k2 > 0) {                                       // per-block summaries beside the accumulated ones

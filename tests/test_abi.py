@@ -47,7 +47,7 @@ def test_workspace_sizes_and_layout(mb):
 
 @pytest.mark.parametrize("kw,code", [
     (dict(D=96), -2), (dict(m=2000), -1), (dict(N=1001), -1), (dict(Cq=0), -1), (dict(k2=9), -2), (dict(k2=1, dtype="f32"), -2),
-    (dict(dipole=1, k2=1), -2), (dict(dipole=2), -1), (dict(Hq=3, Hkv=2), -1), (dict(m=65, Ck=128), -2), (dict(Ck=8192, N=16384), -2),
+    (dict(dipole=1, k2=1), -2), (dict(dipole=3), -1), (dict(Hq=3, Hkv=2), -1), (dict(m=65, Ck=128), -2), (dict(Ck=8192, N=16384), -2),
 ])
 def test_invalid_parameters_are_rejected_on_the_host(mb, kw, code):
     args = dict(B=1, Hq=2, Hkv=2, N=1024, D=64, Cq=8, Ck=16, m=4)

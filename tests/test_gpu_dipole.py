@@ -140,3 +140,66 @@ def test_dipole_backward_matches_oracle(name):
         if moved[key] > 4 * t:
             assert rel_err(got, e) < rel_err(got, plain), key
     assert max(moved.values()) > 4 * t or w.dtype != "f32"
+
+
+# ------------------------------------------------------------------ shared covariance tilted at the mean query centroid
+
+TILT_CASES = {
+    "tiny_f32": (CASES["tiny"].with_(m=0), True, True),
+    "tiny_f32_m2": (CASES["tiny"].with_(m=2), True, True),
+    "tiny_f32_m2_frozen": (CASES["tiny"].with_(m=2), True, False),
+    "tiny_f32_m2_noncausal": (CASES["tiny"].with_(m=2), False, True),
+    "gqa_bf16_d64_m6": (CASES["gqa_bf16"].with_(B=1, Hq=4, Hkv=2, m=6), True, True),     # covariances per query head
+    "d128_bf16_m8": (CASES["d128"].with_(m=8), True, True),
+}
+
+
+@pytest.mark.parametrize("name", list(TILT_CASES))
+def test_tilted_dipole_forward_and_backward_match_oracle(name):
+    from paper_2509_10406_b200 import binding as mb
+    w, causal, agg = TILT_CASES[name]
+    c = Case(w, gain=128.0)
+    qbar32 = c.qbar.astype(np.float32)
+    p = c.params(dipole=2, causal=causal, agg_grad=agg)
+    buf = mb.MuseBuffers(p, backward=True)
+    Q, K, V, dO = c.dev()
+    aq, qb = to_dev(c.a_q, "i"), to_dev(qbar32, "f32")
+    mb.muse_dipole_tilt_point(p, aq, qb, buf.summaries)
+    mb.muse_summarize(p, K, V, to_dev(c.a_k, "i"), qb, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
+    mb.muse_attn_fwd(p, Q, K, V, aq, qb, buf.off_k, buf.perm_k, buf.summaries, None, buf.O, buf.LSE, buf.sel, buf.ws)
+    assert mb.muse_status(buf.ws) == 0
+    mb.muse_attn_bwd(p, Q, K, V, buf.O, buf.LSE, dO, aq, qb, buf.off_k, buf.perm_k, buf.summaries, buf.sel, buf.dQ, buf.dK, buf.dV, buf.ws)
+    torch.cuda.synchronize()
+    assert mb.muse_status(buf.ws) == 0
+    off = mb.muse_dipole_layout(p)
+    qstar = to_np(buf.summaries[off[4]:off[4] + 4 * w.B * w.Hq * w.D].view(torch.float32)).reshape(w.B, w.Hq, w.D)
+    sel = to_np(buf.sel)[..., :w.m]
+    O, dQ, dK, dV = to_np(buf.O), to_np(buf.dQ), to_np(buf.dK), to_np(buf.dV)
+    t = tol(w.dtype)
+    kw = dict(sigma=c.sigma, S=w.S, Ck=w.Ck, m=w.m, causal=causal)
+    far_apart = 0.0
+    for b in range(w.B):
+        for h in range(w.Hq):
+            g = c.hm[h]
+            q64 = qbar32[b, h].astype(np.float64)
+            np.testing.assert_allclose(qstar[b, h], orc.mean_query_centroid(q64, c.a_q[b, h]), rtol=1e-5, atol=1e-6)
+            f2 = orc.forward(c.Q[b, h], c.K[b, g], c.V[b, g], c.a_q[b, h], c.a_k[b, g], q64, dipole=2, sel=sel[b, h] if w.m else None, **kw)
+            f1 = orc.forward(c.Q[b, h], c.K[b, g], c.V[b, g], c.a_q[b, h], c.a_k[b, g], q64, dipole=1, sel=sel[b, h] if w.m else None,
+                             summ=f2["summ"], **kw)
+            assert rel_err(O[b, h], f2["O"]) <= t
+            far_apart = max(far_apart, rel_err(f1["O"], f2["O"]))
+            if rel_err(f1["O"], f2["O"]) > 4 * t:
+                assert rel_err(O[b, h], f2["O"]) < rel_err(O[b, h], f1["O"])
+    args = (c.Q.astype(np.float64), c.K.astype(np.float64), c.V.astype(np.float64), c.dO.astype(np.float64), c.a_q, c.a_k,
+            qbar32.astype(np.float64))
+    eQ, eK, eV = orc.layer_backward(*args, dipole=2, sel=sel, agg_grad=agg, **kw)
+    uQ, uK, uV = orc.layer_backward(*args, dipole=1, sel=sel, agg_grad=agg, **kw)
+    errs = dict(dQ=rel_err(dQ, eQ), dK=rel_err(dK, eK), dV=rel_err(dV, eV))
+    moved = dict(dQ=rel_err(uQ, eQ), dK=rel_err(uK, eK), dV=rel_err(uV, eV))
+    print(name, errs, "tilt moves the output by", far_apart, "and the gradients by", moved)
+    assert all(v <= t for v in errs.values()), errs
+    for key, got, e, plain in (("dQ", dQ, eQ, uQ), ("dK", dK, eK, uK), ("dV", dV, eV, uV)):
+        if moved[key] > 4 * t:
+            assert rel_err(got, e) < rel_err(got, plain), key
+    if w.dtype == "f32":
+        assert far_apart > 4 * t and max(moved.values()) > 4 * t
