@@ -88,6 +88,17 @@ def work_model(w: wl.Workload):
         "k_dipole_merge_tc": ("tensor", 2.0 * heads * SB * Cq * Ck * D * D),
         "k_dipole_merge": ("tensor", 2.0 * heads * SB * Cq * Ck * D * D),
         "k_dipole_apply": ("hbm", heads * SB * Cq * D * D * e + heads * nd * (e + 8)),
+        # ... next to retrieval, and its backward: matrix-vector products per (query, slot) pair and per query,
+        # the two dense contractions over the query and key clusters (all FFMA, counted against the tensor peak
+        # of the same contraction), and the covariance backward to the keys
+        "k_dipole_sub": ("tensor", 2.0 * heads * N * m * (S - 1) / S * D * D),
+        "k_dipole_bwd_pairs": ("tensor", 6.0 * heads * N * m * (S - 1) / S * D * D),
+        "k_dipole_bwd_seg": ("tensor", 4.0 * heads * N * (S - 1) / S * D * D),
+        "k_dipole_dcov": ("tensor", 2.0 * heads * SB * Cq * Ck * D * D),
+        "k_dipole_dpw": ("tensor", 2.0 * heads * SB * Cq * Ck * D * D),
+        "k_dipole_cov_bwd": ("hbm", heads * SB * Ck * D * D * 4 + 2 * heads * nd * (e + 8)),
+        # seeded k-means++ start: every draw reads every vector once
+        "k_kmeanspp": ("hbm", float(nd) * e * (heads * (Cq - 1) + kvh * (Ck - 1))),
     }
     return M
 
@@ -300,8 +311,13 @@ def main():
     ap.add_argument("--clustering", default="lloyd", choices=["lloyd", "streaming"],
                     help="lloyd = muse_cluster (the measured path); streaming = the paper's one-pass mini-batch k-means "
                          "with the balanced per-block assignment (muse_cluster_streaming; device-timed line only)")
-    ap.add_argument("--dipole", action="store_true",
-                    help="far field with the dipole correction instead of retrieval (sets m = 0, forward only)")
+    ap.add_argument("--dipole", type=int, nargs="?", const=1, default=0, choices=[0, 1, 2],
+                    help="far field with the dipole correction: 1 untilted, 2 tilted at the mean query centroid; replaces "
+                         "retrieval (m = 0) unless --dipole-with-retrieval is given (device-timed line only)")
+    ap.add_argument("--dipole-with-retrieval", action="store_true", help="keep m > 0 next to the dipole correction")
+    ap.add_argument("--init", default="indices", choices=["indices", "kmeans++"],
+                    help="start points of Lloyd: indices handed in by the harness (the measured path), or the seeded "
+                         "k-means++ draws on the GPU (MUSE_INIT_KMEANSPP)")
     ap.add_argument("--ref-rows", type=int, default=128, help="sampled queries for the oracle timing")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
@@ -314,8 +330,10 @@ def main():
     if args.m is not None:
         w = w.with_(m=args.m)
     if args.dipole:
-        w = w.with_(m=0)
-        args.forward_only = True
+        if not args.dipole_with_retrieval:
+            w = w.with_(m=0)
+        args.no_e2e = True
+        args.no_cpu_baseline = True
     if args.clustering == "streaming":                    # a device-timed comparison line: no staged run, no oracle sample
         args.no_e2e = True
         args.no_cpu_baseline = True
@@ -360,7 +378,8 @@ def main():
         raise SystemExit("head staging needs B == 1 and a group count that divides the KV heads")
     hq, hkv = w.Hq // groups, w.Hkv // groups
     p = mb.make_params(B=w.B, Hq=hq, Hkv=hkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=w.m, n_blocks=w.S,
-                       dtype=w.dtype, kmeans_iters=w.T, dipole=int(args.dipole), k2=args.k2)
+                       dtype=w.dtype, kmeans_iters=w.T, dipole=int(args.dipole), k2=args.k2,
+                       init_mode=mb.MUSE_INIT_KMEANSPP if args.init == "kmeans++" else mb.MUSE_INIT_INDICES, seed=w.seed)
     buf = mb.MuseBuffers(p, backward=not args.forward_only)
     stream_ws = (torch.zeros(mb.muse_stream_workspace_bytes(p), dtype=torch.uint8, device="cuda")
                  if args.clustering == "streaming" else None)
@@ -380,8 +399,12 @@ def main():
             if args.clustering == "streaming":
                 mb.muse_cluster_streaming(p, Qg, Kg, buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, stream_ws, beta=0.9, cap_factor=4.0)
             else:
-                mb.muse_cluster(p, Qg, Kg, init_q[:, qs], init_k[:, ks], buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, buf.ws)
+                kpp = args.init == "kmeans++"
+                mb.muse_cluster(p, Qg, Kg, None if kpp else init_q[:, qs], None if kpp else init_k[:, ks], buf.assign_q, buf.assign_k,
+                                buf.qbar, buf.kcent, buf.ws)
             m_("cluster")
+            if args.dipole == 2:
+                mb.muse_dipole_tilt_point(p, buf.assign_q, buf.qbar, buf.summaries)
             mb.muse_summarize(p, Kg, Vg, buf.assign_k, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
             m_("summarize")
             mb.muse_attn_fwd(p, Qg, Kg, Vg, buf.assign_q, buf.qbar, buf.off_k, buf.perm_k, buf.summaries, None,
