@@ -236,7 +236,7 @@ int muse_kmeanspp_init(const muse_params_t* p, const void* X, int side, int32_t*
   Arena ar(ws);
   ar.take<int32_t>(kStatusWords);
   float* mind2 = ar.take<float>((size_t)problems * d.N);
-  rc = kmeanspp(p->dtype, X, problems, d.N, d.D, C, side, p->seed, mind2, idx_out, stream);
+  rc = kmeanspp(p->dtype, X, problems, d.N, d.D, C, side, p->seed, mind2, idx_out, (int*)ws, stream);
   prof_mark(nullptr, stream);
   return rc;
 }

@@ -398,7 +398,7 @@ static int lloyd_t(const Dims& d, const T* X, int problems, int C, int kind, con
     // the draws borrow two arrays that the iterations only fill later: perm as the running minimum distance
     // [problems, N] fp32, off (at least C + 1 words per problem) as the drawn indices [problems, C]
     int rc = kmeanspp(sizeof(T) == 2 ? MUSE_BF16 : MUSE_F32, X, problems, d.N, D, C, kind, seed, reinterpret_cast<float*>(perm),
-                      off, st);
+                      off, status, st);
     if (rc != MUSE_OK) return rc;
     init_idx = off;
     init_mode = MUSE_INIT_INDICES;

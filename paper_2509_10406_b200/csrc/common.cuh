@@ -156,7 +156,7 @@ size_t lloyd_ws_bytes(const Dims& d, int problems, int C, int kind);
 // the paper's own clustering: one streaming pass (state = totals, counts; n_batches < 0: to the end) and the
 // per-block assignment under a bucket-size cap (factor <= 0: plain nearest centroid)
 int kmeanspp(int dtype, const void* X, int problems, int N, int D, int C, int kind, uint64_t seed, float* mind2,
-             int32_t* idx_out, cudaStream_t st);
+             int32_t* idx_out, int* status, cudaStream_t st);
 int stream_kmeans(const Dims& d, int dtype, const void* X, int problems, int C, int kind, uint64_t seed, float beta,
                   int first_batch, int n_batches, float* totals, float* counts, float* centres, int32_t* assign_stream,
                   int32_t* status, cudaStream_t st);

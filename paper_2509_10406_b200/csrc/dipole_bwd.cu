@@ -233,12 +233,12 @@ k_dipole_bwd_pairs(Dims dm, const T* __restrict__ Q, const float* __restrict__ q
 }
 
 // ---- dCov[j][x] += sum_i P[i][j] dCbar[i][x]   (x over D*D; thread = one x, 16 key clusters per CTA) ---------------
-constexpr int kDcJ = 16, kDcI = 64;
+constexpr int kDcJ = 32, kDcI = 64;
 
 template <class ST>
 __global__ void __launch_bounds__(256)
 k_dipole_dcov(Dims dm, const ST* __restrict__ P, const float* __restrict__ dcbar, float* __restrict__ dcov) {
-  __shared__ float ps[kDcI][kDcJ];
+  __shared__ __align__(16) float ps[kDcI][kDcJ];
   const int DD = dm.D * dm.D;
   const int x = blockIdx.x * 256 + threadIdx.x, j0 = blockIdx.y * kDcJ;
   const size_t pp = blockIdx.z;
@@ -256,7 +256,11 @@ k_dipole_dcov(Dims dm, const ST* __restrict__ P, const float* __restrict__ dcbar
     for (int ii = 0; ii < ni; ++ii) {
       const float c = dcbar[(pp * dm.Cq + i0 + ii) * DD + x];
 #pragma unroll
-      for (int a = 0; a < kDcJ; ++a) acc[a] = fmaf(ps[ii][a], c, acc[a]);
+      for (int a = 0; a < kDcJ; a += 4) {
+        const float4 p4 = *reinterpret_cast<const float4*>(&ps[ii][a]);
+        acc[a] = fmaf(p4.x, c, acc[a]); acc[a + 1] = fmaf(p4.y, c, acc[a + 1]);
+        acc[a + 2] = fmaf(p4.z, c, acc[a + 2]); acc[a + 3] = fmaf(p4.w, c, acc[a + 3]);
+      }
     }
   }
 #pragma unroll
@@ -264,25 +268,29 @@ k_dipole_dcov(Dims dm, const ST* __restrict__ P, const float* __restrict__ dcbar
     if (j0 + a < dm.Ck) dcov[(pp * dm.Ck + j0 + a) * DD + x] += acc[a];
 }
 
-// ---- dP[i][j] += <dCbar_i, Cov_j> + sum of dZ over the segment   (32 x 32 tile per CTA, 2 x 2 per thread) -----------
+// ---- dP[i][j] += <dCbar_i, Cov_j> + sum of dZ over the segment   (64 x 64 tile per CTA, 4 x 4 per thread) -----------
 template <class ST>
 __global__ void __launch_bounds__(256)
 k_dipole_dpw(Dims dm, const float* __restrict__ dcbar, const ST* __restrict__ cov, const float* __restrict__ dzs,
              float* __restrict__ dpw) {
-  __shared__ float as[32][65], bs[32][65];
+  __shared__ float as[64][33], bs[64][33];
   const int DD = dm.D * dm.D;
-  const int j0 = blockIdx.x * 32, i0 = blockIdx.y * 32, tid = threadIdx.x;
+  const int j0 = blockIdx.x * 64, i0 = blockIdx.y * 64, tid = threadIdx.x;
   const int pp = blockIdx.z, pq = pp / dm.SB, pl = pp % dm.SB;
   const int pk = (pq / dm.Hq) * dm.Hkv + dm.hm.g[pq % dm.Hq];
   const int pc = dm.dipole == 2 ? pq : pk;
   const float* ab = dcbar + ((size_t)pp * dm.Cq) * DD;
   const ST* bb = cov + (((size_t)pc * dm.SB + pl) * dm.Ck) * DD;
   const int ty = tid >> 4, tx = tid & 15;
-  float acc[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-  for (int x0 = 0; x0 < DD; x0 += 64) {
+  float acc[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+  for (int x0 = 0; x0 < DD; x0 += 32) {
     __syncthreads();
-    for (int e = tid; e < 32 * 16; e += 256) {
-      const int r = e / 16, c4 = (e % 16) * 4;
+    for (int e = tid; e < 64 * 8; e += 256) {
+      const int r = e / 8, c4 = (e % 8) * 4;
       float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
       if (i0 + r < dm.Cq) a = ld4(ab + (size_t)(i0 + r) * DD + x0 + c4);
       if (j0 + r < dm.Ck) b = ld4(bb + (size_t)(j0 + r) * DD + x0 + c4);
@@ -291,16 +299,20 @@ k_dipole_dpw(Dims dm, const float* __restrict__ dcbar, const ST* __restrict__ co
     }
     __syncthreads();
 #pragma unroll 8
-    for (int x = 0; x < 64; ++x) {
-      const float a0 = as[ty][x], a1 = as[ty + 16][x], b0 = bs[tx][x], b1 = bs[tx + 16][x];
-      acc[0][0] = fmaf(a0, b0, acc[0][0]); acc[0][1] = fmaf(a0, b1, acc[0][1]);
-      acc[1][0] = fmaf(a1, b0, acc[1][0]); acc[1][1] = fmaf(a1, b1, acc[1][1]);
+    for (int x = 0; x < 32; ++x) {
+      float av_[4], bv_[4];
+#pragma unroll
+      for (int a = 0; a < 4; ++a) { av_[a] = as[ty + 16 * a][x]; bv_[a] = bs[tx + 16 * a][x]; }
+#pragma unroll
+      for (int a = 0; a < 4; ++a)
+#pragma unroll
+        for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av_[a], bv_[b], acc[a][b]);
     }
   }
 #pragma unroll
-  for (int a = 0; a < 2; ++a)
+  for (int a = 0; a < 4; ++a)
 #pragma unroll
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < 4; ++b) {
       const int i = i0 + ty + 16 * a, j = j0 + tx + 16 * b;
       if (i < dm.Cq && j < dm.Ck) dpw[((size_t)pp * dm.Cq + i) * dm.Ck + j] += acc[a][b] + dzs[(size_t)pp * dm.Cq + i];
     }
@@ -558,7 +570,7 @@ static int dipole_bwd_pre_t(const Dims& d, const T* Q, const T* dO, const float*
   MUSE_LAUNCH_OK();
   if (d.agg_grad) {
     prof_mark("k_dipole_dpw", st);
-    k_dipole_dpw<ST><<<dim3(cdiv(d.Ck, 32), cdiv(d.Cq, 32), (unsigned)(pq * d.SB)), 256, 0, st>>>(d, w.dcbar, (const ST*)dp.cov, w.dzs, w.dpw);
+    k_dipole_dpw<ST><<<dim3(cdiv(d.Ck, 64), cdiv(d.Cq, 64), (unsigned)(pq * d.SB)), 256, 0, st>>>(d, w.dcbar, (const ST*)dp.cov, w.dzs, w.dpw);
     MUSE_LAUNCH_OK();
   }
   return MUSE_OK;

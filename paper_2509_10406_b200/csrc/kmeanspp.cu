@@ -7,37 +7,88 @@
 //
 // One problem (head, side) = one thread-block cluster of up to 8 CTAs, each owning a contiguous slice of the vectors;
 // the C - 1 draws are sequential, each ends with one candidate per CTA written into every CTA's shared memory and a
-// hardware cluster barrier.  A draw reads every vector once (distance to the newest start point only, the running
-// minimum lives in scratch), so the stage moves (C - 1) N D e bytes per problem and is bound by L2 / HBM bandwidth.
+// hardware cluster barrier.  A draw reads every vector once (distance to the newest start point only; the running
+// minima stay in shared memory when the slice fits, else in scratch), so the stage moves (C - 1) N D e bytes per
+// problem.  At the headline size it does about 24 instructions per vector, which takes as long as the HBM read: the
+// kernel sits between the issue limit and the bandwidth limit.
 #include <cooperative_groups.h>
 
 #include "common.cuh"
 #include "feistel.cuh"
+#include "tc05.cuh"
 
 namespace cg = cooperative_groups;
 
 namespace muse {
 
-constexpr int kPpThreads = 512, kPpCluster = 8, kPpWarps = kPpThreads / 32;
+constexpr int kPpThreads = 256, kPpCluster = 8, kPpWarps = kPpThreads / 32;
 
 __device__ __forceinline__ bool pp_better(float k, int i, float bk, int bi) { return k > bk || (k == bk && i < bi); }
 
-template <class T, int D>
+// contiguous global -> shared bulk copy (16-byte aligned, size a multiple of 16), completion counted on an mbarrier
+__device__ __forceinline__ void pp_bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(tc::smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(tc::smem_u32(bar)) : "memory");
+}
+
+// Every warp streams its own groups of GR consecutive vectors through a private ring of kPpStages shared-memory
+// stages filled by bulk copies (plain loads top out near 25 bytes per clock per SM here, bulk copies do not); the ring
+// keeps running across draws, since every draw reads the same slice in the same order.
+template <class T, int D, int kPpStages, int kPpGroupBytes>
 __global__ void __launch_bounds__(kPpThreads)
 k_kmeanspp(const T* __restrict__ X, int N, int C, uint64_t seed, int kind, float* __restrict__ mind2,
-           int32_t* __restrict__ idx_out) {
+           int32_t* __restrict__ idx_out, int md_shared, int* __restrict__ status) {
   cg::cluster_group cluster = cg::this_cluster();
   const int CS = (int)cluster.num_blocks(), rank = (int)cluster.block_rank();
   const int prob = blockIdx.x / CS, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int EPL = 16 / (int)sizeof(T);      // elements per 16-byte load
+  constexpr int LPR = D / EPL, RPW = 32 / LPR;  // lanes per vector, vectors per warp and load
+  constexpr int GR = (kPpGroupBytes / (D * (int)sizeof(T))) < 32 ? (kPpGroupBytes / (D * (int)sizeof(T))) : 32;   // vectors per group
+  constexpr int GB = GR * D * (int)sizeof(T);   // bytes per stage (<= 8 KB)
+  constexpr int NL = GR / RPW;                  // loads per lane and group
+  extern __shared__ __align__(128) unsigned char pp_smem[];
   __shared__ float cs[D];
-  __shared__ float exk[2][kPpCluster], wk[kPpWarps];
+  __shared__ float exk[2][kPpCluster], wk[kPpWarps], dpark[kPpWarps][32];
   __shared__ int exi[2][kPpCluster], wi[kPpWarps];
+  __shared__ uint64_t full[kPpWarps][kPpStages];
+  unsigned char* ring = pp_smem + (size_t)warp * kPpStages * GB;
+  float* mds = reinterpret_cast<float*>(pp_smem + (size_t)kPpWarps * kPpStages * GB);   // the slice's running minima, when they fit
   const T* Xp = X + (size_t)prob * N * D;
   float* md = mind2 + (size_t)prob * N;
   const uint64_t stream = (uint64_t)prob * 2 + (uint64_t)kind;
   const int per = (N + CS - 1) / CS, lo = rank * per, hi = min(N, lo + per);
-  constexpr int EPL = D / 8;                    // elements per lane: 8 lanes share one vector
-  const int sub = lane & 7, grp = lane >> 3;
+  const int sub = lane % LPR, grp = lane / LPR;
+  // this warp's groups of one draw: group k covers vectors [lo + (k * kPpWarps + warp) * GR, ... + GR)
+  const int ngroups = hi > lo ? (hi - lo + GR - 1) / GR : 0;
+  const int mine = ngroups > warp ? (ngroups - warp + kPpWarps - 1) / kPpWarps : 0;
+  const int total = mine * (C - 1);             // at most (N / 256) * kMaxC: fits
+  // Every CTA walks its slice from a different starting group (the order inside a draw does not matter: the draw is
+  // a maximum with an explicit tie rule).  Without it all CTAs read the same offset of their 2^k-spaced slices at the
+  // same moment, and the copies crowd onto a few memory channels.
+  const int shift = mine > 0 ? (int)((blockIdx.x * 37u + 11u) % (unsigned)mine) : 0;
+  // running positions instead of divisions: kc / sc = group and stage consumed next, ki / si = group and stage filled next
+  int kc = shift, sc = 0, ki = shift, si = 0, issued = 0;
+  uint32_t phase = 0;                           // bit s = parity of stage s's next completion
+  auto issue = [&]() {                          // lane 0: start the copy of the warp's next group
+    const int k = ki, s = si;
+    ki = ki + 1 == mine ? 0 : ki + 1; si = si + 1 == kPpStages ? 0 : si + 1; ++issued;
+    const int t0 = lo + (k * kPpWarps + warp) * GR;
+    const uint32_t bytes = (uint32_t)min(GR, hi - t0) * (uint32_t)(D * sizeof(T));
+    tc::mbar_expect_tx(&full[warp][s], bytes);
+    pp_bulk_load(ring + s * GB, Xp + (size_t)t0 * D, bytes, &full[warp][s]);
+  };
+  if (lane == 0) {
+    for (int s = 0; s < kPpStages; ++s) tc::mbar_init(&full[warp][s], 1);
+    tc::mbar_init_fence();
+  }
+  __syncwarp();
+  if (lane == 0)
+    while (issued < kPpStages - 1 && issued < total) issue();
+  bool ok = true;
+  // Running minima d2: in shared memory when the slice fits beside the ring (md_shared); otherwise in global scratch,
+  // loaded one group ahead -- a load issued and awaited inside one group costs several microseconds per group when the
+  // memory system is saturated by the copies, and halves the kernel's speed
+  float mcur = INFINITY;
   int last = feistel_permute(0, N, seed, stream);
   if (rank == 0 && tid == 0) idx_out[(size_t)prob * C] = last;
   cluster.sync();                               // every CTA of the problem is running before any of them writes into another's shared memory
@@ -46,41 +97,74 @@ k_kmeanspp(const T* __restrict__ X, int N, int C, uint64_t seed, int kind, float
     __syncthreads();
     float cen[EPL];
 #pragma unroll
-    for (int k = 0; k < EPL / 4; ++k) {
-      const float4 v = *reinterpret_cast<const float4*>(&cs[k * 32 + sub * 4]);
-      cen[k * 4] = v.x; cen[k * 4 + 1] = v.y; cen[k * 4 + 2] = v.z; cen[k * 4 + 3] = v.w;
-    }
+    for (int k = 0; k < EPL; ++k) cen[k] = cs[sub * EPL + k];
     const uint64_t key_c = splitmix64(seed ^ (stream << 32) ^ (0xA5ull << 56) ^ (uint64_t)c);
     float bk = -1.f; int bi = 0x7fffffff;
-#pragma unroll 2
-    for (int t0 = lo + warp * 4; t0 < hi; t0 += kPpWarps * 4) {
-      const int t = t0 + grp;
-      float d = 0.f;
-      if (t < hi) {
+    for (int kk = 0; kk < mine && ok; ++kk) {
+      const int s = sc, k = kc;
+      // refill the stage that was read in the previous iteration (its loads have delivered their values: they were
+      // consumed before the __syncwarp that ended that iteration), then wait for this group's bytes
+      if (lane == 0 && issued < total) issue();
+      // the outcome of the bounded wait is made the same for the whole warp before anyone acts on it
+      if (!__all_sync(0xffffffffu, tc::mbar_wait(&full[warp][s], (phase >> s) & 1u) ? 1 : 0)) { ok = false; break; }
+      phase ^= 1u << s;
+      kc = kc + 1 == mine ? 0 : kc + 1; sc = sc + 1 == kPpStages ? 0 : sc + 1;
+      float mnext = INFINITY;
+      if (!md_shared && kk + 1 < mine && c > 1) {
+        const int tn = lo + (kc * kPpWarps + warp) * GR + lane;
+        if (lane < GR && tn < hi) mnext = md[tn];
+      }
+      const unsigned char* st = ring + s * GB;
+      const int w0 = lo + (k * kPpWarps + warp) * GR;
 #pragma unroll
-        for (int k = 0; k < EPL / 4; ++k) {
-          const float4 v = ld4(Xp + (size_t)t * D + k * 32 + sub * 4);
-          const float a = v.x - cen[k * 4], b = v.y - cen[k * 4 + 1], e = v.z - cen[k * 4 + 2], f = v.w - cen[k * 4 + 3];
-          d = fmaf(a, a, d); d = fmaf(b, b, d); d = fmaf(e, e, d); d = fmaf(f, f, d);
+      for (int h = 0; h < NL; h += 8) {
+        uint4 raw[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          if (h + u < NL) raw[u] = *reinterpret_cast<const uint4*>(st + ((size_t)((h + u) * RPW + grp) * D + sub * EPL) * sizeof(T));
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          if (h + u >= NL) continue;
+          float x[EPL];
+          if (sizeof(T) == 2) {
+            const uint32_t wv[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { x[2 * e] = __uint_as_float(wv[e] << 16); x[2 * e + 1] = __uint_as_float(wv[e] & 0xffff0000u); }
+          } else {
+            x[0] = __uint_as_float(raw[u].x); x[1] = __uint_as_float(raw[u].y);
+            x[EPL - 2] = __uint_as_float(raw[u].z); x[EPL - 1] = __uint_as_float(raw[u].w);
+          }
+          float d = 0.f;
+#pragma unroll
+          for (int e = 0; e < EPL; ++e) { const float a = x[e] - cen[e]; d = fmaf(a, a, d); }
+#pragma unroll
+          for (int o = LPR / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+          if (sub == 0) dpark[warp][(h + u) * RPW + grp] = d;
         }
       }
-      d += __shfl_xor_sync(0xffffffffu, d, 1);
-      d += __shfl_xor_sync(0xffffffffu, d, 2);
-      d += __shfl_xor_sync(0xffffffffu, d, 4);
-      if (sub == 0 && t < hi) {
-        if (c > 1) d = fminf(d, md[t]);
-        md[t] = d;
+      __syncwarp();
+      const int t = w0 + lane;
+      if (lane < GR && t < hi) {                // rows past the slice's end hold stale bytes: never looked at
+        float d = dpark[warp][lane];
+        if (md_shared) { if (c > 1) d = fminf(d, mds[t - lo]); mds[t - lo] = d; }
+        else { d = fminf(d, mcur); md[t] = d; }
         const uint64_t h = splitmix64(key_c ^ (uint64_t)t);
         const float u = ((float)(uint32_t)(h >> 41) + 0.5f) * (1.f / 8388608.f);
         const float key = d / -logf(u);
         if (pp_better(key, t, bk, bi)) { bk = key; bi = t; }
       }
+      __syncwarp();
+      mcur = mnext;
+    }
+    if (!md_shared && mine > 0 && ok) {         // first group of the next draw (this lane wrote its value during this draw)
+      const int tn = lo + (kc * kPpWarps + warp) * GR + lane;
+      mcur = lane < GR && tn < hi ? md[tn] : INFINITY;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-      const float ok = __shfl_xor_sync(0xffffffffu, bk, o);
+      const float ok_ = __shfl_xor_sync(0xffffffffu, bk, o);
       const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (pp_better(ok, oi, bk, bi)) { bk = ok; bi = oi; }
+      if (pp_better(ok_, oi, bk, bi)) { bk = ok_; bi = oi; }
     }
     if (lane == 0) { wk[warp] = bk; wi[warp] = bi; }
     __syncthreads();
@@ -89,9 +173,9 @@ k_kmeanspp(const T* __restrict__ X, int N, int C, uint64_t seed, int kind, float
       bk = lane < kPpWarps ? wk[lane] : -1.f; bi = lane < kPpWarps ? wi[lane] : 0x7fffffff;
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) {
-        const float ok = __shfl_xor_sync(0xffffffffu, bk, o);
+        const float ok_ = __shfl_xor_sync(0xffffffffu, bk, o);
         const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-        if (pp_better(ok, oi, bk, bi)) { bk = ok; bi = oi; }
+        if (pp_better(ok_, oi, bk, bi)) { bk = ok_; bi = oi; }
       }
       if (lane < CS) {                          // lane r delivers this CTA's candidate to CTA r
         *cluster.map_shared_rank(&exk[par][rank], lane) = bk;
@@ -102,8 +186,15 @@ k_kmeanspp(const T* __restrict__ X, int N, int C, uint64_t seed, int kind, float
     bk = -1.f; bi = 0x7fffffff;
     for (int r = 0; r < CS; ++r)
       if (pp_better(exk[par][r], exi[par][r], bk, bi)) { bk = exk[par][r]; bi = exi[par][r]; }
-    last = bi;
+    last = min(max(bi, 0), N - 1);
     if (rank == 0 && tid == 0) idx_out[(size_t)prob * C + c] = last;
+  }
+  if (!ok) {
+    // a wait gave up: say so, and let the (at most kPpStages - 1) copies still in flight land before the CTA's
+    // shared memory is released
+    if (lane == 0) report_status(status, MUSE_STATUS_ASSIGN_TIMEOUT);
+    const long long t0 = clock64();
+    while (clock64() - t0 < (1ll << 24)) { }
   }
   cluster.sync();                               // no CTA leaves while another may still write into its shared memory
 }
@@ -111,37 +202,75 @@ k_kmeanspp(const T* __restrict__ X, int N, int C, uint64_t seed, int kind, float
 size_t kmeanspp_ws_floats(int problems, int N) { return (size_t)problems * N; }
 
 template <class T, int D>
-static int kmeanspp_t(const T* X, int problems, int N, int C, int kind, uint64_t seed, float* mind2, int32_t* idx_out,
-                      cudaStream_t st) {
+struct PpPlan { int stages; int md_shared; size_t smem; };
+
+// Ring depth and where the running minima live for a slice of `per` vectors: three stages when the minima then still
+// fit in shared memory (or do not fit either way), two stages when that is what makes them fit.
+template <class T, int D>
+static PpPlan<T, D> pp_plan(int per) {
+  constexpr int GR = (8192 / (D * (int)sizeof(T))) < 32 ? (8192 / (D * (int)sizeof(T))) : 32;
+  const size_t stage = (size_t)kPpWarps * GR * D * sizeof(T), md_bytes = (size_t)per * sizeof(float), budget = 224 * 1024;
+  if (3 * stage + md_bytes <= budget) return {3, 1, 3 * stage + md_bytes};
+  if (2 * stage + md_bytes <= budget) return {2, 1, 2 * stage + md_bytes};
+  return {3, 0, 3 * stage};
+}
+
+template <class T, int D, int ST>
+static int kmeanspp_v(const T* X, int problems, int N, int C, int kind, uint64_t seed, float* mind2, int32_t* idx_out,
+                      int cs, int md_shared, size_t smem, bool query_only, int* max_clusters, int* status, cudaStream_t st) {
   cudaLaunchConfig_t cfg = {};
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   cfg.stream = st;
-  // CTAs per problem: as many as keep a slice of at least 1024 vectors, up to 8
-  int cs = 1;
-  while (cs < kPpCluster && N >= 2048 * cs) cs *= 2;
   cfg.gridDim = dim3(problems * cs);
   cfg.blockDim = dim3(kPpThreads);
-  cfg.dynamicSmemBytes = 0;
-  attr[0].val.clusterDim.x = cs;
+  cfg.dynamicSmemBytes = smem;
+  MUSE_CUDA_OK(cudaFuncSetAttribute(k_kmeanspp<T, D, ST, 8192>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  if (query_only) {
+    MUSE_CUDA_OK(cudaOccupancyMaxActiveClusters(max_clusters, k_kmeanspp<T, D, ST, 8192>, &cfg));
+    return MUSE_OK;
+  }
   prof_mark("k_kmeanspp", st);
-  MUSE_CUDA_OK(cudaLaunchKernelEx(&cfg, k_kmeanspp<T, D>, X, N, C, seed, kind, mind2, idx_out));
+  MUSE_CUDA_OK(cudaLaunchKernelEx(&cfg, k_kmeanspp<T, D, ST, 8192>, X, N, C, seed, kind, mind2, idx_out, md_shared, status));
   return MUSE_OK;
+}
+
+template <class T, int D>
+static int kmeanspp_t(const T* X, int problems, int N, int C, int kind, uint64_t seed, float* mind2, int32_t* idx_out,
+                      int* status, cudaStream_t st) {
+  // CTAs per problem: the most (up to 8, slices of at least 1024 vectors) for which all problems' clusters can be resident
+  // at once.  The draws are sequential, so a cluster that has to wait for a free slot doubles the stage's time; a GPU
+  // whose processor groups leave no room for every cluster of 8 does better with clusters of 7 or 6.
+  int cs_max = 1;
+  while (cs_max < kPpCluster && N >= 1024 * (cs_max + 1)) ++cs_max;
+  int cs = cs_max;
+  for (int c = cs_max; c >= 1; --c) {
+    const PpPlan<T, D> pl = pp_plan<T, D>((N + c - 1) / c);
+    int active = 0;
+    int rc = pl.stages == 3 ? kmeanspp_v<T, D, 3>(X, problems, N, C, kind, seed, mind2, idx_out, c, pl.md_shared, pl.smem, true, &active, status, st)
+                            : kmeanspp_v<T, D, 2>(X, problems, N, C, kind, seed, mind2, idx_out, c, pl.md_shared, pl.smem, true, &active, status, st);
+    if (rc != MUSE_OK) return rc;
+    if (active >= problems) { cs = c; break; }
+    if (c == 1 || active * c < 64) { cs = cs_max; break; }       // more problems than the GPU holds: several rounds either way
+  }
+  const PpPlan<T, D> pl = pp_plan<T, D>((N + cs - 1) / cs);
+  if (pl.stages == 3) return kmeanspp_v<T, D, 3>(X, problems, N, C, kind, seed, mind2, idx_out, cs, pl.md_shared, pl.smem, false, nullptr, status, st);
+  return kmeanspp_v<T, D, 2>(X, problems, N, C, kind, seed, mind2, idx_out, cs, pl.md_shared, pl.smem, false, nullptr, status, st);
 }
 
 // Start indices [problems, C] of every problem; mind2 is scratch of kmeanspp_ws_floats(problems, N) floats.
 int kmeanspp(int dtype, const void* X, int problems, int N, int D, int C, int kind, uint64_t seed, float* mind2,
-             int32_t* idx_out, cudaStream_t st) {
+             int32_t* idx_out, int* status, cudaStream_t st) {
   typedef __nv_bfloat16 bf;
   if (dtype == MUSE_F32) {
-    if (D == 64) return kmeanspp_t<float, 64>((const float*)X, problems, N, C, kind, seed, mind2, idx_out, st);
-    return kmeanspp_t<float, 128>((const float*)X, problems, N, C, kind, seed, mind2, idx_out, st);
+    if (D == 64) return kmeanspp_t<float, 64>((const float*)X, problems, N, C, kind, seed, mind2, idx_out, status, st);
+    return kmeanspp_t<float, 128>((const float*)X, problems, N, C, kind, seed, mind2, idx_out, status, st);
   }
-  if (D == 64) return kmeanspp_t<bf, 64>((const bf*)X, problems, N, C, kind, seed, mind2, idx_out, st);
-  return kmeanspp_t<bf, 128>((const bf*)X, problems, N, C, kind, seed, mind2, idx_out, st);
+  if (D == 64) return kmeanspp_t<bf, 64>((const bf*)X, problems, N, C, kind, seed, mind2, idx_out, status, st);
+  return kmeanspp_t<bf, 128>((const bf*)X, problems, N, C, kind, seed, mind2, idx_out, status, st);
 }
 
 }  // namespace muse
