@@ -206,16 +206,19 @@ inline SummPtrs summ_ptrs_blk(const SummLayout& L, const void* base_) {      // 
 // dipole correction (dipole.cu): construction at summary time, consumption after the far field
 size_t dipole_fwd_ws_bytes(const Dims& d);
 // its backward (dipole_bwd.cu); scratch carved from the backward workspace
-struct DipoleBwdWs { int32_t* sel_tmp; float *lse_far, *zq, *dz, *delta_far, *xq, *corr, *csub, *dcbar, *dcov, *dpw, *dzs; };
-DipoleBwdWs dipole_bwd_ws(const Dims& d, Arena& ar);
+struct DipoleBwdWs { int32_t* sel_tmp; float *lse_far, *zq, *dz, *delta_far, *xq, *corr, *csub, *dcbar, *dcov, *dpw, *dzs; void* dcbar_bf; };
+DipoleBwdWs dipole_bwd_ws(const Dims& d, Arena& ar);       // sized for either kind of contraction kernel
 bool dipole_bwd_supported(const Dims& d);
+bool dipole_bwd_tc_supported(const Dims& d, int dtype);
+int dipole_bwd_tc(const Dims& d, const void* P, const void* cov, const float* dcbar, void* dcbar_bf, const float* dzs, float* dcov,
+                  float* dpw, int with_dpw, int* status, cudaStream_t st);
 int dipole_tilt_point(const Dims& d, const int32_t* assign_q, const float* qbar, float* qstar, cudaStream_t st);
 int far_fwd_again(const Dims& d, int dtype, const void* Q, const float* qbar, const int32_t* off_q, const int32_t* perm_q,
                   const SummPtrs& sp, const int32_t* sel_in, int32_t* sel_tmp, float* o_far, float* lse_far, int* status,
                   cudaStream_t st);
 int dipole_bwd_pre(const Dims& d, int dtype, const void* Q, const void* dO, const float* qbar, const float* LSE, const float* delta,
                    const int32_t* assign_q, const int32_t* off_q, const int32_t* perm_q, const DipolePtrs& dp, const int32_t* goff,
-                   const int32_t* pairs, const DipoleBwdWs& w, float* dQacc, cudaStream_t st);
+                   const int32_t* pairs, const DipoleBwdWs& w, float* dQacc, int* status, cudaStream_t st);
 int dipole_bwd_dmu(const Dims& d, int dtype, const DipolePtrs& dp, const DipoleBwdWs& w, float* dS, int grad_by_key_cluster,
                    cudaStream_t st);
 int dipole_bwd_keys(const Dims& d, int dtype, const void* Kp, const void* Vp, const int32_t* off_k, const DipolePtrs& dp,

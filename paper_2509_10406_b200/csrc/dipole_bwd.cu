@@ -233,7 +233,7 @@ k_dipole_bwd_pairs(Dims dm, const T* __restrict__ Q, const float* __restrict__ q
 }
 
 // ---- dCov[j][x] += sum_i P[i][j] dCbar[i][x]   (x over D*D; thread = one x, 16 key clusters per CTA) ---------------
-constexpr int kDcJ = 32, kDcI = 64;
+constexpr int kDcJ = 16, kDcI = 64;
 
 template <class ST>
 __global__ void __launch_bounds__(256)
@@ -519,6 +519,7 @@ DipoleBwdWs dipole_bwd_ws(const Dims& d, Arena& ar) {
   w.dcov = ar.take<float>(pq * d.SB * d.Ck * d.D * d.D);
   w.dpw = ar.take<float>(segs * d.Ck);
   w.dzs = ar.take<float>(segs);
+  w.dcbar_bf = ar.take<__nv_bfloat16>(segs * d.D * d.D);      // bf16 copy of dCbar for the tensor-core contractions
   return w;
 }
 
@@ -532,7 +533,8 @@ bool dipole_bwd_supported(const Dims& d) {
 template <class T, class ST, int D>
 static int dipole_bwd_pre_t(const Dims& d, const T* Q, const T* dO, const float* qbar, const float* LSE, const float* delta,
                             const int32_t* assign_q, const int32_t* off_q, const int32_t* perm_q, const DipolePtrs& dp,
-                            const int32_t* goff, const int32_t* pairs, const DipoleBwdWs& w, float* dQacc, cudaStream_t st) {
+                            const int32_t* goff, const int32_t* pairs, const DipoleBwdWs& w, float* dQacc, int* status,
+                            cudaStream_t st) {
   const size_t pq = (size_t)d.B * d.Hq, segs = pq * d.SB * d.Cq;
   const long long rows = (long long)pq * d.N;
   prof_mark("k_dipole_bwd_prep", st);
@@ -565,6 +567,8 @@ static int dipole_bwd_pre_t(const Dims& d, const T* Q, const T* dO, const float*
     prof_mark("memset", st);
     MUSE_CUDA_OK(cudaMemsetAsync(w.dcov, 0, pq * d.SB * d.Ck * D * D * sizeof(float), st));
   }
+  if (dipole_bwd_tc_supported(d, sizeof(ST) == 2 ? MUSE_BF16 : MUSE_F32) && !path_forced(kForceDipoleSimt))
+    return dipole_bwd_tc(d, dp.pw, dp.cov, w.dcbar, w.dcbar_bf, w.dzs, w.dcov, w.dpw, d.agg_grad, status, st);
   prof_mark("k_dipole_dcov", st);
   k_dipole_dcov<ST><<<dim3(D * D / 256, cdiv(d.Ck, kDcJ), (unsigned)(pq * d.SB)), 256, 0, st>>>(d, (const ST*)dp.pw, w.dcbar, w.dcov);
   MUSE_LAUNCH_OK();
@@ -578,9 +582,9 @@ static int dipole_bwd_pre_t(const Dims& d, const T* Q, const T* dO, const float*
 
 int dipole_bwd_pre(const Dims& d, int dtype, const void* Q, const void* dO, const float* qbar, const float* LSE, const float* delta,
                    const int32_t* assign_q, const int32_t* off_q, const int32_t* perm_q, const DipolePtrs& dp, const int32_t* goff,
-                   const int32_t* pairs, const DipoleBwdWs& w, float* dQacc, cudaStream_t st) {
+                   const int32_t* pairs, const DipoleBwdWs& w, float* dQacc, int* status, cudaStream_t st) {
   typedef __nv_bfloat16 bf;
-#define MUSE_DB(TT, SS, DD) dipole_bwd_pre_t<TT, SS, DD>(d, (const TT*)Q, (const TT*)dO, qbar, LSE, delta, assign_q, off_q, perm_q, dp, goff, pairs, w, dQacc, st)
+#define MUSE_DB(TT, SS, DD) dipole_bwd_pre_t<TT, SS, DD>(d, (const TT*)Q, (const TT*)dO, qbar, LSE, delta, assign_q, off_q, perm_q, dp, goff, pairs, w, dQacc, status, st)
   if (dtype == MUSE_F32) return d.D == 64 ? MUSE_DB(float, float, 64) : MUSE_DB(float, float, 128);
   return d.D == 64 ? MUSE_DB(bf, bf, 64) : MUSE_DB(bf, bf, 128);
 #undef MUSE_DB

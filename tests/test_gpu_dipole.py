@@ -7,7 +7,7 @@ import pytest
 import torch
 
 from oracle import muse_oracle as orc
-from tests.gpu_util import Case, to_dev, to_np, tol, rel_err
+from tests.gpu_util import Case, to_dev, to_np, tol, rel_err, kernels_launched
 from tests.test_gpu_cluster import CASES
 
 pytestmark = pytest.mark.gpu
@@ -103,13 +103,35 @@ BWD_CASES = {
     "gqa_bf16_d64_m6": (CASES["gqa_bf16"].with_(B=1, Hq=4, Hkv=2, m=6), True, True),
     "d128_bf16_m8": (CASES["d128"].with_(m=8), True, True),                             # tensor-core far field and key-side pass
     "d128_f32_odd_ck_m5": (CASES["d128"].with_(dtype="f32", m=5, Hq=1, Hkv=1, N=1000, Cq=8, Ck=24, S=4), True, True),
+    # C_q a multiple of 64: the two dense contractions of the backward run on the tensor cores
+    "d128_bf16_tc_m4": (CASES["d128"].with_(Hq=1, Hkv=1, N=1024, Cq=64, Ck=128, m=4, S=4), True, True),
+    "d64_bf16_tc_ragged_ck": (CASES["gqa_bf16"].with_(B=1, Hq=2, Hkv=1, N=1024, Cq=128, Ck=72, m=3, S=4), True, True),
 }
+TC_DIPOLE_BWD = {"k_dipole_dcov_tc", "k_dipole_dpw_tc"}
 
 
 @pytest.mark.parametrize("name", list(BWD_CASES))
 def test_dipole_backward_matches_oracle(name):
     from paper_2509_10406_b200 import binding as mb
     w, causal, agg = BWD_CASES[name]
+    with kernels_launched() as rec:
+        _dipole_backward_case(mb, name, w, causal, agg)
+    assert ("_tc_" in name) == TC_DIPOLE_BWD.issubset(rec.names), sorted(rec.names)
+
+
+def test_dipole_backward_contractions_on_the_plain_kernels_at_a_tensor_shape():
+    from paper_2509_10406_b200 import binding as mb
+    w, causal, agg = BWD_CASES["d64_bf16_tc_ragged_ck"]
+    mb.muse_test_force_paths(mb.FORCE_DIPOLE_SIMT)
+    try:
+        with kernels_launched() as rec:
+            _dipole_backward_case(mb, "forced", w, causal, agg)
+    finally:
+        mb.muse_test_force_paths(0)
+    assert {"k_dipole_dcov", "k_dipole_dpw"}.issubset(rec.names) and not (TC_DIPOLE_BWD & rec.names)
+
+
+def _dipole_backward_case(mb, name, w, causal, agg):
     gain = 128.0
     c = Case(w, gain=gain)
     qbar32 = c.qbar.astype(np.float32)
