@@ -96,6 +96,8 @@ def work_model(w: wl.Workload):
         "k_dipole_bwd_seg": ("tensor", 4.0 * heads * N * (S - 1) / S * D * D),
         "k_dipole_dcov": ("tensor", 2.0 * heads * SB * Cq * Ck * D * D),
         "k_dipole_dpw": ("tensor", 2.0 * heads * SB * Cq * Ck * D * D),
+        "k_dipole_dcov_tc": ("tensor", 2.0 * heads * SB * Cq * Ck * D * D),
+        "k_dipole_dpw_tc": ("tensor", 2.0 * heads * SB * Cq * Ck * D * D),
         "k_dipole_cov_bwd": ("hbm", heads * SB * Ck * D * D * 4 + 2 * heads * nd * (e + 8)),
         # seeded k-means++ start: every draw reads every vector once
         "k_kmeanspp": ("hbm", float(nd) * e * (heads * (Cq - 1) + kvh * (Ck - 1))),

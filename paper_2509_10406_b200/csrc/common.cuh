@@ -211,7 +211,7 @@ DipoleBwdWs dipole_bwd_ws(const Dims& d, Arena& ar);       // sized for either k
 bool dipole_bwd_supported(const Dims& d);
 bool dipole_bwd_tc_supported(const Dims& d, int dtype);
 int dipole_bwd_tc(const Dims& d, const void* P, const void* cov, const float* dcbar, void* dcbar_bf, const float* dzs, float* dcov,
-                  float* dpw, int with_dpw, int* status, cudaStream_t st);
+                  float* dpw, int with_dpw, int dcov_has_terms, int* status, cudaStream_t st);
 int dipole_tilt_point(const Dims& d, const int32_t* assign_q, const float* qbar, float* qstar, cudaStream_t st);
 int far_fwd_again(const Dims& d, int dtype, const void* Q, const float* qbar, const int32_t* off_q, const int32_t* perm_q,
                   const SummPtrs& sp, const int32_t* sel_in, int32_t* sel_tmp, float* o_far, float* lse_far, int* status,

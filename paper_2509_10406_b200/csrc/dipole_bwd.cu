@@ -563,12 +563,13 @@ static int dipole_bwd_pre_t(const Dims& d, const T* Q, const T* dO, const float*
     k_dipole_bwd_pairs<T, ST, D><<<dim3(d.Ck, d.SB, (unsigned)pq), 256, smem, st>>>(d, Q, qbar, assign_q, goff, pairs, (const ST*)dp.cov,
                                                                                    (const ST*)dp.pw, w.xq, w.dz, dQacc, w.dcov, w.dpw);
     MUSE_LAUNCH_OK();
-  } else {
+  }
+  const bool tensor = dipole_bwd_tc_supported(d, sizeof(ST) == 2 ? MUSE_BF16 : MUSE_F32) && !path_forced(kForceDipoleSimt);
+  if (d.m == 0 && !tensor) {                              // the plain kernel adds to dCov; the tensor kernel can overwrite it
     prof_mark("memset", st);
     MUSE_CUDA_OK(cudaMemsetAsync(w.dcov, 0, pq * d.SB * d.Ck * D * D * sizeof(float), st));
   }
-  if (dipole_bwd_tc_supported(d, sizeof(ST) == 2 ? MUSE_BF16 : MUSE_F32) && !path_forced(kForceDipoleSimt))
-    return dipole_bwd_tc(d, dp.pw, dp.cov, w.dcbar, w.dcbar_bf, w.dzs, w.dcov, w.dpw, d.agg_grad, status, st);
+  if (tensor) return dipole_bwd_tc(d, dp.pw, dp.cov, w.dcbar, w.dcbar_bf, w.dzs, w.dcov, w.dpw, d.agg_grad, d.m > 0 ? 1 : 0, status, st);
   prof_mark("k_dipole_dcov", st);
   k_dipole_dcov<ST><<<dim3(D * D / 256, cdiv(d.Ck, kDcJ), (unsigned)(pq * d.SB)), 256, 0, st>>>(d, (const ST*)dp.pw, w.dcbar, w.dcov);
   MUSE_LAUNCH_OK();

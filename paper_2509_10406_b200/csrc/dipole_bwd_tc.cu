@@ -35,7 +35,7 @@ __global__ void k_to_bf16(const float* __restrict__ src, size_t n4, bf16* __rest
 template <int MODE>
 __global__ void __launch_bounds__(128)
 k_dipole_bwd_gemm_tc(Dims dm, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                     const float* __restrict__ dzs, float* __restrict__ out, int* __restrict__ status) {
+                     const float* __restrict__ dzs, float* __restrict__ out, int accumulate, int* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ DbBars bars;
   __shared__ uint32_t tbase_s;
@@ -120,12 +120,12 @@ k_dipole_bwd_gemm_tc(Dims dm, const __grid_constant__ CUtensorMap tm_a, const __
       for (int c = 0; c < 32; c += 4) {
         const int col = n0 + 32 * q + c;
         if (col + 3 < cols) {
-          float4 o = *reinterpret_cast<float4*>(orow + 32 * q + c);
+          float4 o = accumulate ? *reinterpret_cast<float4*>(orow + 32 * q + c) : make_float4(0.f, 0.f, 0.f, 0.f);
           o.x += v[c] + add; o.y += v[c + 1] + add; o.z += v[c + 2] + add; o.w += v[c + 3] + add;
           *reinterpret_cast<float4*>(orow + 32 * q + c) = o;
         } else {
           for (int e = 0; e < 4; ++e)
-            if (col + e < cols) orow[32 * q + c + e] += v[c + e] + add;
+            if (col + e < cols) orow[32 * q + c + e] = (accumulate ? orow[32 * q + c + e] : 0.f) + v[c + e] + add;
         }
       }
     }
@@ -144,8 +144,9 @@ bool dipole_bwd_tc_supported(const Dims& d, int dtype) {
 }
 
 // dcbar_bf: scratch for the bf16 copy of dCbar ([B*Hq*SB*Cq][D*D]).
+// dcov_has_terms: dCov already holds the retrieved clusters' (negative) share and is added to; otherwise it is overwritten.
 int dipole_bwd_tc(const Dims& d, const void* P, const void* cov, const float* dcbar, void* dcbar_bf, const float* dzs, float* dcov,
-                  float* dpw, int with_dpw, int* status, cudaStream_t st) {
+                  float* dpw, int with_dpw, int dcov_has_terms, int* status, cudaStream_t st) {
   const int DD = d.D * d.D;
   const uint64_t rows_p = (uint64_t)d.B * d.Hq * d.SB * d.Cq, rows_c = (uint64_t)d.B * (d.dipole == 2 ? d.Hq : d.Hkv) * d.SB * d.Ck;
   const size_t n4 = rows_p * DD / 4;
@@ -162,11 +163,11 @@ int dipole_bwd_tc(const Dims& d, const void* P, const void* cov, const float* dc
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_bwd_gemm_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_bwd_gemm_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prof_mark("k_dipole_dcov_tc", st);
-  k_dipole_bwd_gemm_tc<0><<<dim3(DD / 128, cdiv(d.Ck, 128), d.B * d.Hq * d.SB), 128, smem, st>>>(d, tp64, tg64, nullptr, dcov, status);
+  k_dipole_bwd_gemm_tc<0><<<dim3(DD / 128, cdiv(d.Ck, 128), d.B * d.Hq * d.SB), 128, smem, st>>>(d, tp64, tg64, nullptr, dcov, dcov_has_terms, status);
   MUSE_LAUNCH_OK();
   if (with_dpw) {
     prof_mark("k_dipole_dpw_tc", st);
-    k_dipole_bwd_gemm_tc<1><<<dim3(cdiv(d.Ck, 128), cdiv(d.Cq, 128), d.B * d.Hq * d.SB), 128, smem, st>>>(d, tg128, tc128, dzs, dpw, status);
+    k_dipole_bwd_gemm_tc<1><<<dim3(cdiv(d.Ck, 128), cdiv(d.Cq, 128), d.B * d.Hq * d.SB), 128, smem, st>>>(d, tg128, tc128, dzs, dpw, 1, status);
     MUSE_LAUNCH_OK();
   }
   return MUSE_OK;

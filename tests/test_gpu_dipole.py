@@ -106,6 +106,7 @@ BWD_CASES = {
     # C_q a multiple of 64: the two dense contractions of the backward run on the tensor cores
     "d128_bf16_tc_m4": (CASES["d128"].with_(Hq=1, Hkv=1, N=1024, Cq=64, Ck=128, m=4, S=4), True, True),
     "d64_bf16_tc_ragged_ck": (CASES["gqa_bf16"].with_(B=1, Hq=2, Hkv=1, N=1024, Cq=128, Ck=72, m=3, S=4), True, True),
+    "d64_bf16_tc_m0": (CASES["gqa_bf16"].with_(B=1, Hq=2, Hkv=2, N=1024, Cq=64, Ck=200, m=0, S=4), True, True),
 }
 TC_DIPOLE_BWD = {"k_dipole_dcov_tc", "k_dipole_dpw_tc"}
 
