@@ -200,15 +200,22 @@ __device__ __forceinline__ void load_cov_t(const CT* __restrict__ cb, float* Ct,
   }
 }
 
+// Register tile: a thread owns 4 consecutive value dims of kSubQ pairs; the covariance sits transposed in shared memory
+// in its storage type (Ct[key dim][value dim], rows 16-byte aligned), so that per 4 key dims a thread reads 4 vectors of
+// the matrix and kSubQ broadcast vectors of residuals for 16 * kSubQ multiply-adds -- with one value dim per thread the
+// kernel was bound by shared-memory reads at a fifth of the FMA rate.
+constexpr int kSubQ = 8;
+
 template <class T, class ST, int D>
 __global__ void __launch_bounds__(256)
 k_dipole_sub(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, const int32_t* __restrict__ assign_q,
              const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs, const ST* __restrict__ cov,
              const ST* __restrict__ pw, float* __restrict__ csub) {
-  constexpr int G = 256 / D, R = G * kApplyQ;   // query groups working side by side, pairs per pass
-  extern __shared__ float smd[];
-  float* Ct = smd;
-  float* qs = Ct + D * (D + 1);                 // [R][D] residuals
+  constexpr int TG = D / 4, G = 256 / TG, R = G * kSubQ;      // threads per pair group, groups, pairs per pass
+  constexpr int P = D + 16 / (int)sizeof(ST);                 // pitch of a Ct row (elements)
+  extern __shared__ __align__(16) unsigned char smd_raw[];
+  float* qs = reinterpret_cast<float*>(smd_raw);              // [R][D] residuals
+  ST* Ct = reinterpret_cast<ST*>(qs + R * D);                 // [D key dims][P]
   __shared__ int t_s[R], i_s[R];
   __shared__ float p_s[R];
   const int j = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z, tid = threadIdx.x;
@@ -217,12 +224,13 @@ k_dipole_sub(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, c
   if (g0 >= g1) return;
   const int pk = (pq / dm.Hq) * dm.Hkv + dm.hm.g[pq % dm.Hq];
   const int pc = dm.dipole == 2 ? pq : pk;      // the tilted covariance belongs to a query head
-  load_cov_t<ST, D>(cov + (((size_t)pc * dm.SB + pl) * dm.Ck + j) * D * D, Ct, tid);
+  const ST* cb = cov + (((size_t)pc * dm.SB + pl) * dm.Ck + j) * D * D;
+  for (int e = tid; e < D * D; e += 256) Ct[(e % D) * P + e / D] = cb[e];          // cov[dv][dk] -> Ct[dk][dv]
   const T* Qp = Q + (size_t)pq * dm.N * D;
   const int32_t* aq = assign_q + (size_t)pq * dm.N;
   const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
   const ST* pwb = pw + ((size_t)pq * dm.SB + pl) * dm.Cq * dm.Ck;
-  const int grp = tid / D, dv = tid % D;
+  const int grp = tid / TG, d4 = (tid % TG) * 4;
   for (int r0 = g0; r0 < g1; r0 += R) {
     __syncthreads();
     if (tid < R) {
@@ -236,24 +244,40 @@ k_dipole_sub(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, c
       p_s[tid] = t >= 0 ? to_f(pwb[(size_t)i * dm.Ck + j]) : 0.f;
     }
     __syncthreads();
-    for (int e = tid; e < R * D; e += 256) {
-      const int r = e / D, dk = e % D, t = t_s[r];
-      qs[e] = t >= 0 ? dm.sigma * (to_f(Qp[(size_t)t * D + dk]) - qbar[((size_t)pq * dm.Cq + i_s[r]) * D + dk]) : 0.f;
+    for (int e = tid; e < R * (D / 4); e += 256) {
+      const int r = e / (D / 4), c4 = (e % (D / 4)) * 4, t = t_s[r];
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (t >= 0) {
+        const float4 q = ld4(Qp + (size_t)t * D + c4), b = ld4(qbar + ((size_t)pq * dm.Cq + i_s[r]) * D + c4);
+        v = make_float4(dm.sigma * (q.x - b.x), dm.sigma * (q.y - b.y), dm.sigma * (q.z - b.z), dm.sigma * (q.w - b.w));
+      }
+      st4(qs + r * D + c4, v);
     }
     __syncthreads();
-    float acc[kApplyQ];
+    float acc[kSubQ][4];
 #pragma unroll
-    for (int a = 0; a < kApplyQ; ++a) acc[a] = 0.f;
-    const float* qg = qs + grp * kApplyQ * D;
-    for (int dk = 0; dk < D; ++dk) {
-      const float c = Ct[dk * (D + 1) + dv];
+    for (int a = 0; a < kSubQ; ++a) { acc[a][0] = 0.f; acc[a][1] = 0.f; acc[a][2] = 0.f; acc[a][3] = 0.f; }
+    const float* qg = qs + grp * kSubQ * D;
+#pragma unroll 2
+    for (int dk = 0; dk < D; dk += 4) {
+      const float4 c0 = ld4(Ct + (dk + 0) * P + d4), c1 = ld4(Ct + (dk + 1) * P + d4);
+      const float4 c2 = ld4(Ct + (dk + 2) * P + d4), c3 = ld4(Ct + (dk + 3) * P + d4);
 #pragma unroll
-      for (int a = 0; a < kApplyQ; ++a) acc[a] = fmaf(c, qg[a * D + dk], acc[a]);
+      for (int a = 0; a < kSubQ; ++a) {
+        const float4 q = *reinterpret_cast<const float4*>(qg + a * D + dk);
+        acc[a][0] = fmaf(c0.x, q.x, fmaf(c1.x, q.y, fmaf(c2.x, q.z, fmaf(c3.x, q.w, acc[a][0]))));
+        acc[a][1] = fmaf(c0.y, q.x, fmaf(c1.y, q.y, fmaf(c2.y, q.z, fmaf(c3.y, q.w, acc[a][1]))));
+        acc[a][2] = fmaf(c0.z, q.x, fmaf(c1.z, q.y, fmaf(c2.z, q.z, fmaf(c3.z, q.w, acc[a][2]))));
+        acc[a][3] = fmaf(c0.w, q.x, fmaf(c1.w, q.y, fmaf(c2.w, q.z, fmaf(c3.w, q.w, acc[a][3]))));
+      }
     }
 #pragma unroll
-    for (int a = 0; a < kApplyQ; ++a) {
-      const int r = grp * kApplyQ + a, t = t_s[r];
-      if (t >= 0) atomicAdd(&csub[((size_t)pq * dm.N + t) * D + dv], p_s[r] * acc[a]);
+    for (int a = 0; a < kSubQ; ++a) {
+      const int r = grp * kSubQ + a, t = t_s[r];
+      const float p = p_s[r];
+      if (t >= 0)
+        atomicAdd(reinterpret_cast<float4*>(&csub[((size_t)pq * dm.N + t) * D + d4]),
+                  make_float4(p * acc[a][0], p * acc[a][1], p * acc[a][2], p * acc[a][3]));
     }
   }
 }
@@ -305,12 +329,7 @@ k_dipole_apply(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar,
     float acc[kApplyQ];
 #pragma unroll
     for (int a = 0; a < kApplyQ; ++a) acc[a] = 0.f;
-    const float* qg = qs + grp * kApplyQ * D;
-    for (int dk = 0; dk < D; ++dk) {
-      const float c = Ct[dk * (D + 1) + dv];
-#pragma unroll
-      for (int a = 0; a < kApplyQ; ++a) acc[a] = fmaf(c, qg[a * D + dk], acc[a]);
-    }
+    matvec_rows<D, kApplyQ>(Ct, qs + grp * kApplyQ * D, dv, acc);
 #pragma unroll
     for (int a = 0; a < kApplyQ; ++a) {
       const int r = r0 + grp * kApplyQ + a;
@@ -406,10 +425,11 @@ static int dipole_apply_t(const Dims& d, const T* Q, const float* qbar, const in
   const size_t smem = (size_t)(D * (D + 1) + (256 / D) * kApplyQ * D) * sizeof(float);
   const dim3 grid(d.Cq, d.SB, d.B * d.Hq);
   if (d.m > 0) {
+    const size_t ssub = (size_t)(256 / (D / 4)) * kSubQ * D * sizeof(float) + (size_t)D * (D + 16 / sizeof(ST)) * sizeof(ST);
     MUSE_CUDA_OK(cudaMemsetAsync(csub, 0, (size_t)d.B * d.Hq * d.N * D * sizeof(float), st));
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_sub<T, ST, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_sub<T, ST, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssub));
     prof_mark("k_dipole_sub", st);
-    k_dipole_sub<T, ST, D><<<dim3(d.Ck, d.SB, d.B * d.Hq), 256, smem, st>>>(d, Q, qbar, assign_q, goff, pairs, (const ST*)dp.cov,
+    k_dipole_sub<T, ST, D><<<dim3(d.Ck, d.SB, d.B * d.Hq), 256, ssub, st>>>(d, Q, qbar, assign_q, goff, pairs, (const ST*)dp.cov,
                                                                             (const ST*)dp.pw, csub);
     MUSE_LAUNCH_OK();
     if (sizeof(ST) == 2) {

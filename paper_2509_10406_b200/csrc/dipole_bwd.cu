@@ -106,11 +106,16 @@ k_dipole_bwd_seg(Dims dm, const T* __restrict__ Q, const float* __restrict__ qba
     float acc[kDbQ];
 #pragma unroll
     for (int a = 0; a < kDbQ; ++a) acc[a] = 0.f;
+    // Ct is indexed [dk][dv] here and the sum runs over dv: the untransposed product, read along a row of Ct
     const float* xg = xs + grp * kDbQ * D;
-    for (int dv = 0; dv < D; ++dv) {
-      const float c = Ct[dk * (D + 1) + dv];
+#pragma unroll 2
+    for (int dv = 0; dv < D; dv += 4) {
+      const float c0 = Ct[dk * (D + 1) + dv], c1 = Ct[dk * (D + 1) + dv + 1], c2 = Ct[dk * (D + 1) + dv + 2], c3 = Ct[dk * (D + 1) + dv + 3];
 #pragma unroll
-      for (int a = 0; a < kDbQ; ++a) acc[a] = fmaf(c, xg[a * D + dv], acc[a]);
+      for (int a = 0; a < kDbQ; ++a) {
+        const float4 x = *reinterpret_cast<const float4*>(xg + a * D + dv);
+        acc[a] = fmaf(c0, x.x, acc[a]); acc[a] = fmaf(c1, x.y, acc[a]); acc[a] = fmaf(c2, x.z, acc[a]); acc[a] = fmaf(c3, x.w, acc[a]);
+      }
     }
 #pragma unroll
     for (int a = 0; a < kDbQ; ++a) {
@@ -144,31 +149,44 @@ k_dipole_bwd_seg(Dims dm, const T* __restrict__ Q, const float* __restrict__ qba
 }
 
 // ---- per (key cluster j, plane, head) group of the inverse index: what the retrieved clusters take back -----------
+// The covariance sits in shared memory as stored ([value dim][key dim], rows 16-byte aligned); a thread owns 4 consecutive
+// key dims of kPairQ pairs for v = Cov^T x (4 matrix vectors + kPairQ broadcast vectors per 16 * kPairQ multiply-adds),
+// and a TV x TV block of the group's outer-product sum.
+constexpr int kPairQ = 8;
+
 template <class T, class ST, int D>
 __global__ void __launch_bounds__(256)
 k_dipole_bwd_pairs(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, const int32_t* __restrict__ assign_q,
                    const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs, const ST* __restrict__ cov,
                    const ST* __restrict__ pw, const float* __restrict__ xq, const float* __restrict__ dz,
                    float* __restrict__ dQacc, float* __restrict__ dcov, float* __restrict__ dpw) {
-  constexpr int G = 256 / D, R = G * kDbQ, TV = D / 16;
-  extern __shared__ float smd[];
-  float* Ct = smd;
-  float* qs = Ct + D * (D + 1);
-  float* xs = qs + R * D;
+  constexpr int TG = D / 4, G = 256 / TG, R = G * kPairQ, TV = D / 16;
+  constexpr int P = D + 16 / (int)sizeof(ST);
+  extern __shared__ __align__(16) unsigned char smd_raw[];
+  float* qs = reinterpret_cast<float*>(smd_raw);              // [R][D] residuals
+  float* xs = qs + R * D;                                     // [R][D] x rows
+  ST* Cs = reinterpret_cast<ST*>(xs + R * D);                 // [D value dims][P]
   __shared__ int t_s[R], i_s[R];
   __shared__ float p_s[R], s_s[R];
-  const int j = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z, tid = threadIdx.x, lane = tid & 31;
+  const int j = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z, tid = threadIdx.x;
   const int32_t* go = goff + (size_t)pq * (dm.SB * dm.Ck + 1) + (size_t)j * dm.SB + pl;
   const int g0 = go[0], g1 = go[1];
   const int pk = (pq / dm.Hq) * dm.Hkv + dm.hm.g[pq % dm.Hq];
   const int pc = dm.dipole == 2 ? pq : pk;
-  const int grp = tid / D, dk = tid % D, ty = tid >> 4, tx = tid & 15;
+  const int grp = tid / TG, d4 = (tid % TG) * 4, ty = tid >> 4, tx = tid & 15;
   float A[TV][TV];
 #pragma unroll
   for (int a = 0; a < TV; ++a)
 #pragma unroll
     for (int c = 0; c < TV; ++c) A[a][c] = 0.f;
-  if (g0 < g1) db_load_t<ST, D>(cov + (((size_t)pc * dm.SB + pl) * dm.Ck + j) * D * D, Ct, tid, 1.f);
+  if (g0 < g1) {
+    const ST* cb = cov + (((size_t)pc * dm.SB + pl) * dm.Ck + j) * D * D;
+    constexpr int V = 16 / (int)sizeof(ST);                   // elements per 16-byte copy
+    for (int e = tid; e < D * D / V; e += 256) {
+      const int dv = e / (D / V), c = (e % (D / V)) * V;
+      *reinterpret_cast<uint4*>(Cs + dv * P + c) = *reinterpret_cast<const uint4*>(cb + (size_t)dv * D + c);
+    }
+  }
   const T* Qp = Q + (size_t)pq * dm.N * D;
   const int32_t* aq = assign_q + (size_t)pq * dm.N;
   const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
@@ -182,32 +200,51 @@ k_dipole_bwd_pairs(Dims dm, const T* __restrict__ Q, const float* __restrict__ q
         if (!MUSE_IN_RANGE(t, dm.N)) t = -1;
       }
       if (t >= 0) { i = aq[t]; if (!MUSE_IN_RANGE(i, dm.Cq)) { t = -1; i = 0; } }
-      t_s[tid] = t; i_s[tid] = i; s_s[tid] = 0.f;
+      t_s[tid] = t; i_s[tid] = i;
       p_s[tid] = t >= 0 ? to_f(pw[(prow + i) * dm.Ck + j]) : 0.f;
     }
     __syncthreads();
-    for (int e = tid; e < R * D; e += 256) {
-      const int r = e / D, c = e % D, t = t_s[r];
-      qs[e] = t >= 0 ? dm.sigma * (to_f(Qp[(size_t)t * D + c]) - qbar[((size_t)pq * dm.Cq + i_s[r]) * D + c]) : 0.f;
-      xs[e] = t >= 0 ? xq[((size_t)pq * dm.N + t) * D + c] : 0.f;
+    for (int e = tid; e < R * (D / 4); e += 256) {
+      const int r = e / (D / 4), c4 = (e % (D / 4)) * 4, t = t_s[r];
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f), x = v;
+      if (t >= 0) {
+        const float4 q = ld4(Qp + (size_t)t * D + c4), b = ld4(qbar + ((size_t)pq * dm.Cq + i_s[r]) * D + c4);
+        v = make_float4(dm.sigma * (q.x - b.x), dm.sigma * (q.y - b.y), dm.sigma * (q.z - b.z), dm.sigma * (q.w - b.w));
+        x = ld4(xq + ((size_t)pq * dm.N + t) * D + c4);
+      }
+      st4(qs + r * D + c4, v); st4(xs + r * D + c4, x);
     }
     __syncthreads();
     // v[dk] = sum_dv Cov[dv][dk] x[dv]:  dqres -= p v,  x^T Cov qres = v . qres
-    float acc[kDbQ];
+    float acc[kPairQ][4];
 #pragma unroll
-    for (int a = 0; a < kDbQ; ++a) acc[a] = 0.f;
-    const float* xg = xs + grp * kDbQ * D;
-    for (int dv = 0; dv < D; ++dv) {
-      const float c = Ct[dk * (D + 1) + dv];
+    for (int a = 0; a < kPairQ; ++a) { acc[a][0] = 0.f; acc[a][1] = 0.f; acc[a][2] = 0.f; acc[a][3] = 0.f; }
+    const float* xg = xs + grp * kPairQ * D;
+#pragma unroll 2
+    for (int dv = 0; dv < D; dv += 4) {
+      const float4 c0 = ld4(Cs + (dv + 0) * P + d4), c1 = ld4(Cs + (dv + 1) * P + d4);
+      const float4 c2 = ld4(Cs + (dv + 2) * P + d4), c3 = ld4(Cs + (dv + 3) * P + d4);
 #pragma unroll
-      for (int a = 0; a < kDbQ; ++a) acc[a] = fmaf(c, xg[a * D + dv], acc[a]);
+      for (int a = 0; a < kPairQ; ++a) {
+        const float4 x = *reinterpret_cast<const float4*>(xg + a * D + dv);
+        acc[a][0] = fmaf(c0.x, x.x, fmaf(c1.x, x.y, fmaf(c2.x, x.z, fmaf(c3.x, x.w, acc[a][0]))));
+        acc[a][1] = fmaf(c0.y, x.x, fmaf(c1.y, x.y, fmaf(c2.y, x.z, fmaf(c3.y, x.w, acc[a][1]))));
+        acc[a][2] = fmaf(c0.z, x.x, fmaf(c1.z, x.y, fmaf(c2.z, x.z, fmaf(c3.z, x.w, acc[a][2]))));
+        acc[a][3] = fmaf(c0.w, x.x, fmaf(c1.w, x.y, fmaf(c2.w, x.z, fmaf(c3.w, x.w, acc[a][3]))));
+      }
     }
 #pragma unroll
-    for (int a = 0; a < kDbQ; ++a) {
-      const int r = grp * kDbQ + a, t = t_s[r];
-      const float part = warp_sum(acc[a] * qs[r * D + dk]);
-      if (lane == 0) atomicAdd(&s_s[r], part);
-      if (t >= 0) atomicAdd(&dQacc[((size_t)pq * dm.N + t) * D + dk], -dm.sigma * p_s[r] * acc[a]);
+    for (int a = 0; a < kPairQ; ++a) {
+      const int r = grp * kPairQ + a, t = t_s[r];
+      const float4 q = *reinterpret_cast<const float4*>(qs + r * D + d4);
+      float part = acc[a][0] * q.x + acc[a][1] * q.y + acc[a][2] * q.z + acc[a][3] * q.w;
+#pragma unroll
+      for (int o = TG / 2; o > 0; o >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o);
+      if (tid % TG == 0) s_s[r] = part;
+      const float f = -dm.sigma * p_s[r];
+      if (t >= 0)
+        atomicAdd(reinterpret_cast<float4*>(&dQacc[((size_t)pq * dm.N + t) * D + d4]),
+                  make_float4(f * acc[a][0], f * acc[a][1], f * acc[a][2], f * acc[a][3]));
     }
     for (int r = 0; r < R; ++r) {
       const float p = p_s[r];
@@ -558,9 +595,10 @@ static int dipole_bwd_pre_t(const Dims& d, const T* Q, const T* dO, const float*
   }
   MUSE_LAUNCH_OK();
   if (d.m > 0) {
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_bwd_pairs<T, ST, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const size_t spair = (size_t)2 * (256 / (D / 4)) * kPairQ * D * sizeof(float) + (size_t)D * (D + 16 / sizeof(ST)) * sizeof(ST);
+    MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_bwd_pairs<T, ST, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)spair));
     prof_mark("k_dipole_bwd_pairs", st);
-    k_dipole_bwd_pairs<T, ST, D><<<dim3(d.Ck, d.SB, (unsigned)pq), 256, smem, st>>>(d, Q, qbar, assign_q, goff, pairs, (const ST*)dp.cov,
+    k_dipole_bwd_pairs<T, ST, D><<<dim3(d.Ck, d.SB, (unsigned)pq), 256, spair, st>>>(d, Q, qbar, assign_q, goff, pairs, (const ST*)dp.cov,
                                                                                    (const ST*)dp.pw, w.xq, w.dz, dQacc, w.dcov, w.dpw);
     MUSE_LAUNCH_OK();
   }
