@@ -430,23 +430,31 @@ k_dipole_cov_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, co
     __syncthreads();
   }
   const float lmax = lmax_s;
-  // prefix means per plane (plane pl = blocks 0..pl), weighted by f_u
-  if (tid < 2 * D) {
+  // prefix means per plane (plane pl = blocks 0..pl), weighted by f_u; with the tilt the weights of eight keys at a
+  // time are computed by the eight warps (one dot product each) and shared
+  {
     const bool isv = tid >= D;
     const int c = tid % D;
     float s = 0.f, wsum = 0.f;
     for (int pl = 0; pl < dm.SB; ++pl) {
-      for (int u = off[pl]; u < off[pl + 1]; ++u) {
-        float f = 1.f;
-        if (TILT) {                             // every thread recomputes the key's weight (a cluster has few keys)
-          float l = 0.f;
-          for (int cc = 0; cc < D; ++cc) l = fmaf(qs_[cc], to_f(Kb[(size_t)u * D + cc]) - k0[cc], l);
-          f = expf(l - lmax);
+      if (TILT) {
+        for (int u0 = off[pl]; u0 < off[pl + 1]; u0 += 8) {
+          const int nk = min(8, off[pl + 1] - u0);
+          const float l = warp < nk ? logit(u0 + warp) : 0.f;
+          if (lane == 0) fk[warp] = warp < nk ? expf(l - lmax) : 0.f;
+          __syncthreads();
+          if (tid < 2 * D)
+            for (int r = 0; r < nk; ++r) {
+              s = fmaf(fk[r], isv ? to_f(Vb[(size_t)(u0 + r) * D + c]) : to_f(Kb[(size_t)(u0 + r) * D + c]) - k0[c], s);
+              wsum += fk[r];
+            }
+          __syncthreads();
         }
-        s = fmaf(f, isv ? to_f(Vb[(size_t)u * D + c]) : to_f(Kb[(size_t)u * D + c]) - k0[c], s);
-        wsum += f;
+      } else if (tid < 2 * D) {
+        for (int u = off[pl]; u < off[pl + 1]; ++u) s += isv ? to_f(Vb[(size_t)u * D + c]) : to_f(Kb[(size_t)u * D + c]) - k0[c];
+        wsum = (float)(off[pl + 1] - first);
       }
-      (isv ? vb : kb)[pl * D + c] = wsum > 0.f ? s / wsum : 0.f;
+      if (tid < 2 * D) (isv ? vb : kb)[pl * D + c] = wsum > 0.f ? s / wsum : 0.f;
       if (tid == 0) wb[pl] = wsum;
     }
   }
