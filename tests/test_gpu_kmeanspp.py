@@ -96,3 +96,40 @@ def test_kmeanspp_start_spreads_over_separated_blobs():
     got = to_np(idx)[0]
     assert sorted(lab[got].tolist()) == list(range(C))
     np.testing.assert_array_equal(got, orc.kmeanspp_init(X.astype(np.float64), C, 5, 0))
+
+
+def test_kmeanspp_full_size_sampled_draws():
+    """Headline shapes, all 16 heads and both sides in one call each (the launch configuration `bench.py --init kmeans++`
+    times): every head's indices are distinct and in range; for one head and side, sampled draws are checked against the
+    oracle, which recomputes the draw from the GPU's earlier start points."""
+    import bench
+    mb = _mb()
+    w = wl.WORKLOADS["headline"]
+    Qh, Kh, _, _, _, _ = bench.gen_inputs(w, 1.0)
+    p = mb.make_params(B=w.B, Hq=w.Hq, Hkv=w.Hkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=w.m, n_blocks=w.S, dtype=w.dtype, seed=w.seed)
+    ws = torch.zeros(mb.muse_workspace_bytes(p)[0], dtype=torch.uint8, device="cuda")
+    got = {}
+    for side, Xh, H, C in ((0, Qh, w.Hq, w.Cq), (1, Kh, w.Hkv, w.Ck)):
+        X = torch.from_numpy(Xh).to(torch.bfloat16).cuda()
+        idx = torch.full((w.B * H, C), -1, dtype=torch.int32, device="cuda")
+        mb.muse_kmeanspp_init(p, X, side, idx, ws)
+        torch.cuda.synchronize()
+        assert mb.muse_status(ws) == 0
+        got[side] = to_np(idx)
+        for pr in range(w.B * H):
+            assert len(set(got[side][pr].tolist())) == C and got[side][pr].min() >= 0 and got[side][pr].max() < w.N
+            assert got[side][pr, 0] == orc.feistel_permute(0, w.N, w.seed, pr * 2 + side)
+    h, side = 5, 1
+    X = Kh[0, h].astype(np.float64)                              # bf16-exact values
+    xn = (X * X).sum(1)
+    picks = got[side][h]
+    near = 0
+    for c in (1, 2, 17, 100, 333, 512, 800, 1023):
+        cen = X[picks[:c]]
+        d2 = np.maximum(xn[:, None] + (cen * cen).sum(1)[None, :] - 2.0 * (X @ cen.T), 0.0).min(1)
+        d2[picks[:c]] = 0.0
+        want, keys = orc.kmeanspp_step(d2, c, w.seed, h * 2 + side)
+        if picks[c] != want:
+            assert keys[picks[c]] >= keys[want] * (1 - 1e-5), (c, picks[c], want)
+            near += 1
+    assert near <= 1
