@@ -99,3 +99,44 @@ def test_headline_shaped_head_elementwise_gradients():
                 dV=rel_err(to_np(buf.dV), eV))
     print("headline-shaped head, N = 16384:", errs)
     assert all(v <= 2e-2 for v in errs.values()), errs
+
+
+def test_headline_full_size_tilted_dipole_next_to_retrieval_sampled_parity():
+    """The dipole options at the benchmark's full size and launch configuration (`bench.py --dipole 2
+    --dipole-with-retrieval`): shared covariance tilted at the mean query centroid, correction restricted to the clusters a
+    query did not retrieve, forward and backward.  O, LSE and dQ of sampled queries of one head against the oracle with the
+    GPU's assignments, centroids and selections; the sum identities on all heads (the correction has zero total weight:
+    it moves values, not mass)."""
+    import bench
+    from paper_2509_10406_b200 import binding as mb
+    w = wl.WORKLOADS["headline"]
+    Qh, Kh, Vh, dOh, iq, ik = bench.gen_inputs(w, 128.0)
+    dev = lambda a: torch.from_numpy(a).to(torch.bfloat16).cuda()
+    Q, K, V, dO = dev(Qh), dev(Kh), dev(Vh), dev(dOh)
+    p = mb.make_params(B=w.B, Hq=w.Hq, Hkv=w.Hkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=w.m, n_blocks=w.S, dtype=w.dtype,
+                       kmeans_iters=w.T, dipole=2)
+    buf = mb.MuseBuffers(p, backward=True)
+    mb.muse_layer_forward(p, buf, Q, K, V, torch.from_numpy(iq).cuda(), torch.from_numpy(ik).cuda())
+    mb.muse_layer_backward(p, buf, Q, K, V, dO)
+    torch.cuda.synchronize()
+    assert mb.muse_status(buf.ws) == 0
+    h = 3
+    a_q, a_k = to_np(buf.assign_q[0, h]), to_np(buf.assign_k[0, h])
+    qbar = to_np(buf.qbar[0, h]).astype(np.float64)
+    rng = np.random.default_rng(1)
+    rows = np.sort(np.concatenate([rng.choice(np.arange(b * 8192, (b + 1) * 8192), 2, replace=False) for b in range(8)]))
+    sel = to_np(buf.sel[0, h])
+    Q64, K64, V64, dO64 = (x[0, h].astype(np.float64) for x in (Qh, Kh, Vh, dOh))
+    kw = dict(sigma=1.0 / np.sqrt(w.D), S=w.S, Ck=w.Ck, m=w.m, sel=sel, rows=rows)
+    dQ, _, _, f = orc.backward(Q64, K64, V64, dO64, a_q, a_k, qbar, dipole=2, **kw)
+    plain = orc.forward(Q64, K64, V64, a_q, a_k, qbar, **kw)
+    O, LSE, gQ = to_np(buf.O[0, h]), to_np(buf.LSE[0, h]), to_np(buf.dQ[0, h])
+    errs = dict(O=rel_err(O[rows], f["O"][rows]), LSE=float(np.abs(LSE[rows] - f["LSE"][rows]).max() / np.abs(f["LSE"][rows]).max()),
+                dQ=rel_err(gQ[rows], dQ[rows]))
+    moved = rel_err(plain["O"][rows], f["O"][rows])
+    print("full-size tilted dipole next to retrieval (head %d, %d queries):" % (h, rows.size), errs, "correction moves O by", moved)
+    assert all(v <= 2e-2 for v in errs.values()), errs
+    dV, dK = buf.dV.float(), buf.dK.float()
+    sum_dO = dO.float().sum(2)
+    assert float((dV.sum(2) - sum_dO).abs().max() / sum_dO.abs().max()) <= 2e-2
+    assert float(dK.sum(2).abs().max() / dK.abs().sum(2).max()) <= 2e-2
