@@ -687,8 +687,9 @@ def main():
         context["sharp_inputs_device_status"] = mb.muse_status(buf.ws)
         Q.mul_(1.0 / 128.0)
     if not args.no_sharp and args.clustering == "lloyd" and args.k2 == 0 and not args.dipole and w.dtype == "bf16" and groups == 1:
-        # the path's two options on the same inputs, device-timed, as context beside the headline numbers: the paper's own
-        # clustering in place of Lloyd (cluster stage only), and the two-level retrieval with k2 = 1 (summarize + forward)
+        # the path's options on the same inputs, device-timed, as context beside the headline numbers: the paper's own
+        # clustering in place of Lloyd and Lloyd from the k-means++ start drawn on the GPU (cluster stage only), the two-level
+        # retrieval with k2 = 1 and the dipole correction with m = 0 (summarize + forward)
         try:
             sws = torch.zeros(mb.muse_stream_workspace_bytes(p), dtype=torch.uint8, device="cuda")
             for it in range(3):
@@ -699,6 +700,15 @@ def main():
             context["streaming_clustering_stage_ms"] = ev0.elapsed_time(ev1) / 2
             context["streaming_clustering_device_status"] = mb.muse_status(sws)
             del sws
+            pk = mb.make_params(B=w.B, Hq=hq, Hkv=hkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=w.m, n_blocks=w.S, dtype=w.dtype,
+                                kmeans_iters=w.T, init_mode=mb.MUSE_INIT_KMEANSPP, seed=w.seed)
+            for it in range(3):
+                if it == 1:
+                    ev0.record()
+                mb.muse_cluster(pk, Q, K, None, None, buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, buf.ws)
+            ev1.record(); torch.cuda.synchronize()
+            context["kmeanspp_start_clustering_stage_ms"] = ev0.elapsed_time(ev1) / 2
+            context["kmeanspp_start_device_status"] = mb.muse_status(buf.ws)
             mb.muse_cluster(p, Q, K, init_q, init_k, buf.assign_q, buf.assign_k, buf.qbar, buf.kcent, buf.ws)
             p2 = mb.make_params(B=w.B, Hq=hq, Hkv=hkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=w.m, n_blocks=w.S, dtype=w.dtype,
                                 kmeans_iters=w.T, k2=1)
@@ -719,6 +729,20 @@ def main():
                 context["k2_all_summarize_plus_forward_ms"] = stages.get("summarize", 0.0) + stages.get("forward", 0.0)
                 context["two_level_device_status"] = mb.muse_status(b2.ws)
                 del b2
+                torch.cuda.empty_cache()
+                # the dipole correction as the paper defines it (no retrieval): summarize + forward
+                p3 = mb.make_params(B=w.B, Hq=hq, Hkv=hkv, N=w.N, D=w.D, Cq=w.Cq, Ck=w.Ck, m=0, n_blocks=w.S, dtype=w.dtype,
+                                    kmeans_iters=w.T, dipole=1)
+                b3 = mb.MuseBuffers(p3, backward=False)
+                for it in range(3):
+                    if it == 1:
+                        ev0.record()
+                    mb.muse_summarize(p3, K, V, ak, qb, b3.off_k, b3.perm_k, b3.summaries, b3.ws)
+                    mb.muse_attn_fwd(p3, Q, K, V, aq, qb, b3.off_k, b3.perm_k, b3.summaries, None, O_all, b3.LSE, b3.sel, b3.ws)
+                ev1.record(); torch.cuda.synchronize()
+                context["dipole_m0_summarize_plus_forward_ms"] = ev0.elapsed_time(ev1) / 2
+                context["dipole_device_status"] = mb.muse_status(b3.ws)
+                del b3
         except Exception as ex:
             context["options_error"] = repr(ex)[:200]
     context["paper"] = ("2x over cuDNN flash attention at 64k and +36% pretraining throughput, 8xA100, "
