@@ -107,6 +107,9 @@ BWD_CASES = {
     "d128_bf16_tc_m4": (CASES["d128"].with_(Hq=1, Hkv=1, N=1024, Cq=64, Ck=128, m=4, S=4), True, True),
     "d64_bf16_tc_ragged_ck": (CASES["gqa_bf16"].with_(B=1, Hq=2, Hkv=1, N=1024, Cq=128, Ck=72, m=3, S=4), True, True),
     "d64_bf16_tc_m0": (CASES["gqa_bf16"].with_(B=1, Hq=2, Hkv=2, N=1024, Cq=64, Ck=200, m=0, S=4), True, True),
+    # odd sizes everywhere, three query heads per kv head, two batches
+    "odd_f32_gqa3": (CASES["tiny"].with_(name="odd3", B=2, Hq=3, Hkv=1, N=720, S=3, Cq=5, Ck=13, m=3, components=16), True, True),
+    "odd_f32_d128_noncausal": (CASES["d128"].with_(name="odd128", dtype="f32", Hq=2, Hkv=2, N=516, S=2, Cq=3, Ck=7, m=2, components=8), False, True),
 }
 TC_DIPOLE_BWD = {"k_dipole_dcov_tc", "k_dipole_dpw_tc"}
 
@@ -174,6 +177,8 @@ TILT_CASES = {
     "tiny_f32_m2_noncausal": (CASES["tiny"].with_(m=2), False, True),
     "gqa_bf16_d64_m6": (CASES["gqa_bf16"].with_(B=1, Hq=4, Hkv=2, m=6), True, True),     # covariances per query head
     "d128_bf16_m8": (CASES["d128"].with_(m=8), True, True),
+    "odd_f32_gqa3": (CASES["tiny"].with_(name="odd3", B=2, Hq=3, Hkv=1, N=720, S=3, Cq=5, Ck=13, m=3, components=16), True, True),
+    "odd_bf16_d128_m0": (CASES["d128"].with_(name="odd128", Hq=2, Hkv=2, N=516, S=2, Cq=3, Ck=7, m=0, components=8), True, False),
 }
 
 
