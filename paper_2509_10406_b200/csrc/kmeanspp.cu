@@ -9,9 +9,10 @@
 // the C - 1 draws are sequential, each ends with one candidate per CTA written into every CTA's shared memory and a
 // hardware cluster barrier.  A draw reads every vector once (distance to the newest start point only; the running
 // minima stay in shared memory when the slice fits, else in scratch), so the stage moves (C - 1) N D e bytes per
-// problem.  At the headline size it does about 24 instructions per vector, which takes as long as the HBM read: the
+// problem.  At the headline size its instructions per vector take about as long as the HBM read: the
 // kernel sits between the issue limit and the bandwidth limit.
 #include <cooperative_groups.h>
+#include <type_traits>
 
 #include "common.cuh"
 #include "feistel.cuh"
@@ -61,7 +62,8 @@ k_kmeanspp(const T* __restrict__ X, int N, int C, uint64_t seed, int kind, float
   // this warp's groups of one draw: group k covers vectors [lo + (k * kPpWarps + warp) * GR, ... + GR)
   const int ngroups = hi > lo ? (hi - lo + GR - 1) / GR : 0;
   const int mine = ngroups > warp ? (ngroups - warp + kPpWarps - 1) / kPpWarps : 0;
-  const int total = mine * (C - 1);             // at most (N / 256) * kMaxC: fits
+  const bool norms = md_shared != 0 && C > 1;   // squared norms kept beside the minima: the cheaper distance form
+  const int total = mine * (C - 1 + (norms ? 1 : 0));      // at most (N / 256) * (kMaxC + 1): fits
   // Every CTA walks its slice from a different starting group (the order inside a draw does not matter: the draw is
   // a maximum with an explicit tie rule).  Without it all CTAs read the same offset of their 2^k-spaced slices at the
   // same moment, and the copies crowd onto a few memory channels.
@@ -85,67 +87,73 @@ k_kmeanspp(const T* __restrict__ X, int N, int C, uint64_t seed, int kind, float
   if (lane == 0)
     while (issued < kPpStages - 1 && issued < total) issue();
   bool ok = true;
-  // Running minima d2: in shared memory when the slice fits beside the ring (md_shared); otherwise in global scratch,
-  // loaded one group ahead -- a load issued and awaited inside one group costs several microseconds per group when the
-  // memory system is saturated by the copies, and halves the kernel's speed
+  // Running minima d2 (and, with them, the squared norms): in shared memory when the slice fits beside the ring
+  // (md_shared); otherwise the minima live in global scratch and are loaded one group ahead.
+  float* xns = mds + per;                       // squared norms of the slice's vectors (md_shared only)
   float mcur = INFINITY;
+  float cen[EPL];
+  float cn = 0.f;                               // squared norm of the newest start point
+  uint64_t key_c = 0;
+  float bk = -1.f; int bi = 0x7fffffff;
   int last = feistel_permute(0, N, seed, stream);
-  if (rank == 0 && tid == 0) idx_out[(size_t)prob * C] = last;
-  cluster.sync();                               // every CTA of the problem is running before any of them writes into another's shared memory
-  for (int c = 1; c < C; ++c) {
-    if (tid < D) cs[tid] = MUSE_IN_RANGE(last, N) ? to_f(Xp[(size_t)last * D + tid]) : 0.f;
-    __syncthreads();
-    float cen[EPL];
+  // One group of the warp: refill the ring, wait for the group's bytes, reduce every vector against `cen`, finish one
+  // vector per lane.  MODE 0: squared norms (once, before the first draw); MODE 1: draw with d2 = sum (x - c)^2;
+  // MODE 2: draw with d2 = |x|^2 + |c|^2 - 2 x.c from the stored norms (a third fewer instructions per element; the
+  // cancellation error, about 1e-7 of |x|^2 + |c|^2, is far below what separates the race's leaders).
+  auto consume = [&](auto mode_tag, int c, bool more_in_pass) -> bool {
+    constexpr int MODE = decltype(mode_tag)::value;
+    const int s = sc, k = kc;
+    // (the stage read in the previous iteration is free: its loads delivered their values before that iteration's
+    // closing __syncwarp)
+    if (lane == 0 && issued < total) issue();
+    // the outcome of the bounded wait is made the same for the whole warp before anyone acts on it
+    if (!__all_sync(0xffffffffu, tc::mbar_wait(&full[warp][s], (phase >> s) & 1u) ? 1 : 0)) return false;
+    phase ^= 1u << s;
+    kc = kc + 1 == mine ? 0 : kc + 1; sc = sc + 1 == kPpStages ? 0 : sc + 1;
+    float mnext = INFINITY;
+    if (MODE != 0 && !md_shared && more_in_pass && c > 1) {
+      const int tn = lo + (kc * kPpWarps + warp) * GR + lane;
+      if (lane < GR && tn < hi) mnext = md[tn];
+    }
+    const unsigned char* st = ring + s * GB;
+    const int w0 = lo + (k * kPpWarps + warp) * GR;
 #pragma unroll
-    for (int k = 0; k < EPL; ++k) cen[k] = cs[sub * EPL + k];
-    const uint64_t key_c = splitmix64(seed ^ (stream << 32) ^ (0xA5ull << 56) ^ (uint64_t)c);
-    float bk = -1.f; int bi = 0x7fffffff;
-    for (int kk = 0; kk < mine && ok; ++kk) {
-      const int s = sc, k = kc;
-      // refill the stage that was read in the previous iteration (its loads have delivered their values: they were
-      // consumed before the __syncwarp that ended that iteration), then wait for this group's bytes
-      if (lane == 0 && issued < total) issue();
-      // the outcome of the bounded wait is made the same for the whole warp before anyone acts on it
-      if (!__all_sync(0xffffffffu, tc::mbar_wait(&full[warp][s], (phase >> s) & 1u) ? 1 : 0)) { ok = false; break; }
-      phase ^= 1u << s;
-      kc = kc + 1 == mine ? 0 : kc + 1; sc = sc + 1 == kPpStages ? 0 : sc + 1;
-      float mnext = INFINITY;
-      if (!md_shared && kk + 1 < mine && c > 1) {
-        const int tn = lo + (kc * kPpWarps + warp) * GR + lane;
-        if (lane < GR && tn < hi) mnext = md[tn];
-      }
-      const unsigned char* st = ring + s * GB;
-      const int w0 = lo + (k * kPpWarps + warp) * GR;
+    for (int h = 0; h < NL; h += 8) {
+      uint4 raw[8];
 #pragma unroll
-      for (int h = 0; h < NL; h += 8) {
-        uint4 raw[8];
+      for (int u = 0; u < 8; ++u)
+        if (h + u < NL) raw[u] = *reinterpret_cast<const uint4*>(st + ((size_t)((h + u) * RPW + grp) * D + sub * EPL) * sizeof(T));
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-          if (h + u < NL) raw[u] = *reinterpret_cast<const uint4*>(st + ((size_t)((h + u) * RPW + grp) * D + sub * EPL) * sizeof(T));
+      for (int u = 0; u < 8; ++u) {
+        if (h + u >= NL) continue;
+        float x[EPL];
+        if (sizeof(T) == 2) {
+          const uint32_t wv[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          if (h + u >= NL) continue;
-          float x[EPL];
-          if (sizeof(T) == 2) {
-            const uint32_t wv[4] = {raw[u].x, raw[u].y, raw[u].z, raw[u].w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) { x[2 * e] = __uint_as_float(wv[e] << 16); x[2 * e + 1] = __uint_as_float(wv[e] & 0xffff0000u); }
-          } else {
-            x[0] = __uint_as_float(raw[u].x); x[1] = __uint_as_float(raw[u].y);
-            x[EPL - 2] = __uint_as_float(raw[u].z); x[EPL - 1] = __uint_as_float(raw[u].w);
-          }
-          float d = 0.f;
-#pragma unroll
-          for (int e = 0; e < EPL; ++e) { const float a = x[e] - cen[e]; d = fmaf(a, a, d); }
-#pragma unroll
-          for (int o = LPR / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
-          if (sub == 0) dpark[warp][(h + u) * RPW + grp] = d;
+          for (int e = 0; e < 4; ++e) { x[2 * e] = __uint_as_float(wv[e] << 16); x[2 * e + 1] = __uint_as_float(wv[e] & 0xffff0000u); }
+        } else {
+          x[0] = __uint_as_float(raw[u].x); x[1] = __uint_as_float(raw[u].y);
+          x[EPL - 2] = __uint_as_float(raw[u].z); x[EPL - 1] = __uint_as_float(raw[u].w);
         }
+        float d = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+          if (MODE == 0) d = fmaf(x[e], x[e], d);
+          else if (MODE == 1) { const float a = x[e] - cen[e]; d = fmaf(a, a, d); }
+          else d = fmaf(x[e], cen[e], d);
+        }
+#pragma unroll
+        for (int o = LPR / 2; o > 0; o >>= 1) d += __shfl_xor_sync(0xffffffffu, d, o);
+        if (sub == 0) dpark[warp][(h + u) * RPW + grp] = d;
       }
-      __syncwarp();
-      const int t = w0 + lane;
-      if (lane < GR && t < hi) {                // rows past the slice's end hold stale bytes: never looked at
-        float d = dpark[warp][lane];
+    }
+    __syncwarp();
+    const int t = w0 + lane;
+    if (lane < GR && t < hi) {                  // rows past the slice's end hold stale bytes: never looked at
+      float d = dpark[warp][lane];
+      if (MODE == 0) xns[t - lo] = d;
+      else {
+        if (MODE == 2) d = t == last ? 0.f : fmaxf(xns[t - lo] + cn - 2.f * d, 0.f);
         if (md_shared) { if (c > 1) d = fminf(d, mds[t - lo]); mds[t - lo] = d; }
         else { d = fminf(d, mcur); md[t] = d; }
         const uint64_t h = splitmix64(key_c ^ (uint64_t)t);
@@ -153,9 +161,27 @@ k_kmeanspp(const T* __restrict__ X, int N, int C, uint64_t seed, int kind, float
         const float key = d / -logf(u);
         if (pp_better(key, t, bk, bi)) { bk = key; bi = t; }
       }
-      __syncwarp();
-      mcur = mnext;
     }
+    __syncwarp();
+    mcur = mnext;
+    return true;
+  };
+  if (rank == 0 && tid == 0) idx_out[(size_t)prob * C] = last;
+  cluster.sync();                               // every CTA of the problem is running before any of them writes into another's shared memory
+  if (norms)
+    for (int kk = 0; kk < mine && ok; ++kk) ok = consume(std::integral_constant<int, 0>(), 0, kk + 1 < mine);
+  for (int c = 1; c < C; ++c) {
+    if (tid < D) cs[tid] = MUSE_IN_RANGE(last, N) ? to_f(Xp[(size_t)last * D + tid]) : 0.f;
+    __syncthreads();
+    cn = 0.f;
+#pragma unroll
+    for (int k = 0; k < EPL; ++k) { cen[k] = cs[sub * EPL + k]; cn = fmaf(cen[k], cen[k], cn); }
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) cn += __shfl_xor_sync(0xffffffffu, cn, o);
+    key_c = splitmix64(seed ^ (stream << 32) ^ (0xA5ull << 56) ^ (uint64_t)c);
+    bk = -1.f; bi = 0x7fffffff;
+    for (int kk = 0; kk < mine && ok; ++kk)
+      ok = norms ? consume(std::integral_constant<int, 2>(), c, kk + 1 < mine) : consume(std::integral_constant<int, 1>(), c, kk + 1 < mine);
     if (!md_shared && mine > 0 && ok) {         // first group of the next draw (this lane wrote its value during this draw)
       const int tn = lo + (kc * kPpWarps + warp) * GR + lane;
       mcur = lane < GR && tn < hi ? md[tn] : INFINITY;
@@ -209,7 +235,7 @@ struct PpPlan { int stages; int md_shared; size_t smem; };
 template <class T, int D>
 static PpPlan<T, D> pp_plan(int per) {
   constexpr int GR = (8192 / (D * (int)sizeof(T))) < 32 ? (8192 / (D * (int)sizeof(T))) : 32;
-  const size_t stage = (size_t)kPpWarps * GR * D * sizeof(T), md_bytes = (size_t)per * sizeof(float), budget = 224 * 1024;
+  const size_t stage = (size_t)kPpWarps * GR * D * sizeof(T), md_bytes = 2 * (size_t)per * sizeof(float), budget = 224 * 1024;   // minima + norms
   if (3 * stage + md_bytes <= budget) return {3, 1, 3 * stage + md_bytes};
   if (2 * stage + md_bytes <= budget) return {2, 1, 2 * stage + md_bytes};
   return {3, 0, 3 * stage};
