@@ -779,7 +779,7 @@ static int attn_bwd_t(const Dims& d, int dtype, const T* Q, const T* K, const T*
       rc = far_fwd_again(d, dtype, Q, qbar, w.off_q, w.perm_q, sp, sel, w.dip.sel_tmp, w.dip.xq, w.dip.lse_far, w.status, st);
       if (rc != MUSE_OK) return rc;
       rc = dipole_apply(d, dtype, Q, qbar, assign_q, w.off_q, w.perm_q, dp, w.dip.lse_far, sel, ri.goff, ri.pairs, w.dip.csub, nullptr,
-                        w.dip.corr, w.dip.zq, st);
+                        w.dip.corr, w.dip.zq, w.status, st);
       if (rc != MUSE_OK) return rc;
       rc = dipole_bwd_pre(d, dtype, Q, dO, qbar, LSE, w.delta, assign_q, w.off_q, w.perm_q, dp, ri.goff, ri.pairs, w.dip, w.dQacc,
                           w.status, st);

@@ -630,7 +630,7 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
     }
     if (d.dipole && d.m == 0) {
       rc = dipole_apply(d, dtype, Q, qbar, assign_q, w.off_q, w.perm_q, dipole_ptrs(L, base), w.lse_far, nullptr, nullptr, nullptr,
-                        nullptr, w.o_far, nullptr, nullptr, st);
+                        nullptr, w.o_far, nullptr, nullptr, w.status, st);
       if (rc != MUSE_OK) return rc;
     }
     if (d.m > 0) {
@@ -639,7 +639,7 @@ static int attn_fwd_t(const Dims& d, const T* Q, const T* K, const T* V, const i
       if (rc != MUSE_OK) return rc;
       if (d.dipole) {
         rc = dipole_apply(d, dtype, Q, qbar, assign_q, w.off_q, w.perm_q, dipole_ptrs(L, base), w.lse_far, sel, ri.goff, ri.pairs,
-                          w.csub, w.o_far, nullptr, nullptr, st);
+                          w.csub, w.o_far, nullptr, nullptr, w.status, st);
         if (rc != MUSE_OK) return rc;
       }
       if (kTensor) {

@@ -227,7 +227,7 @@ int dipole_build(const Dims& d, int dtype, const void* Kp, const void* Vp, const
                  const DipolePtrs& dp, int* status, cudaStream_t st);
 int dipole_apply(const Dims& d, int dtype, const void* Q, const float* qbar, const int32_t* assign_q, const int32_t* off_q,
                  const int32_t* perm_q, const DipolePtrs& dp, const float* lse_far, const int32_t* sel, const int32_t* goff,
-                 const int32_t* pairs, float* csub, float* o_far, float* corr, float* zq, cudaStream_t st);
+                 const int32_t* pairs, float* csub, float* o_far, float* corr, float* zq, int* status, cudaStream_t st);
 // ST = storage element type of kappa / nu (float or bf16); idx = element index (entry * D + d), d % 4 == 0
 template <class ST> __device__ __forceinline__ float4 ld_kappa4(const SummPtrs& s, size_t idx);
 template <> __device__ __forceinline__ float4 ld_kappa4<float>(const SummPtrs& s, size_t idx) { return ld4((const float*)s.khi + idx); }

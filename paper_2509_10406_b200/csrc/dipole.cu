@@ -21,6 +21,9 @@ namespace muse {
 
 bool dipole_merge_tc_supported(const Dims& d, int dtype);
 int dipole_merge_tc(const Dims& d, const void* P, const void* cov, void* cbar, int out_f32, int* status, cudaStream_t st);
+bool dipole_sub_tc_supported(const Dims& d, int dtype);
+int dipole_sub_tc(const Dims& d, const void* Q, const float* qbar, const int32_t* assign_q, const int32_t* goff, const int32_t* pairs,
+                  const void* cov, const void* pw, float* csub, int* status, cudaStream_t st);
 
 // ---- 1. untilted accumulated covariance ------------------------------------------------------
 // One CTA per (key cluster j, kv head): walks the cluster's buckets in block order with running
@@ -290,7 +293,7 @@ __global__ void __launch_bounds__(256)
 k_dipole_apply(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, const int32_t* __restrict__ off_q,
                const int32_t* __restrict__ perm_q, const CT* __restrict__ cbar, const float* __restrict__ lse_far,
                const int32_t* __restrict__ sel, const ST* __restrict__ pw, const float* __restrict__ zall,
-               const float* __restrict__ csub, float* __restrict__ o_far, float* __restrict__ corr, float* __restrict__ zq) {
+               const float* __restrict__ csub, int round_q, float* __restrict__ o_far, float* __restrict__ corr, float* __restrict__ zq) {
   constexpr int G = 256 / D, R = G * kApplyQ;
   extern __shared__ float smd[];
   float* Ct = smd;                              // [D key dims][D + 1]: transposed matrix, value dim fastest
@@ -323,7 +326,9 @@ k_dipole_apply(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar,
     }
     for (int e = tid; e < R * D; e += 256) {
       const int r = e / D, dk = e % D;
-      qs[e] = r0 + r < p1 ? dm.sigma * (to_f(Qp[(size_t)pm[r0 + r] * D + dk]) - qb[dk]) : 0.f;
+      float v = r0 + r < p1 ? dm.sigma * (to_f(Qp[(size_t)pm[r0 + r] * D + dk]) - qb[dk]) : 0.f;
+      if (round_q) v = __bfloat162float(__float2bfloat16_rn(v));     // the same residuals as the tensor-core kernel that made csub
+      qs[e] = v;
     }
     __syncthreads();
     float acc[kApplyQ];
@@ -421,22 +426,30 @@ template <class T, class ST, int D>
 static int dipole_apply_t(const Dims& d, const T* Q, const float* qbar, const int32_t* assign_q, const int32_t* off_q,
                           const int32_t* perm_q, const DipolePtrs& dp, const float* lse_far, const int32_t* sel,
                           const int32_t* goff, const int32_t* pairs, float* csub, float* o_far, float* corr, float* zq,
-                          cudaStream_t st) {
+                          int* status, cudaStream_t st) {
   const size_t smem = (size_t)(D * (D + 1) + (256 / D) * kApplyQ * D) * sizeof(float);
   const dim3 grid(d.Cq, d.SB, d.B * d.Hq);
+  int round_q = 0;
   if (d.m > 0) {
     const size_t ssub = (size_t)(256 / (D / 4)) * kSubQ * D * sizeof(float) + (size_t)D * (D + 16 / sizeof(ST)) * sizeof(ST);
     MUSE_CUDA_OK(cudaMemsetAsync(csub, 0, (size_t)d.B * d.Hq * d.N * D * sizeof(float), st));
-    MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_sub<T, ST, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssub));
-    prof_mark("k_dipole_sub", st);
-    k_dipole_sub<T, ST, D><<<dim3(d.Ck, d.SB, d.B * d.Hq), 256, ssub, st>>>(d, Q, qbar, assign_q, goff, pairs, (const ST*)dp.cov,
-                                                                            (const ST*)dp.pw, csub);
-    MUSE_LAUNCH_OK();
+    const bool tensor = sizeof(ST) == 2 && dipole_sub_tc_supported(d, MUSE_BF16) && !path_forced(kForceDipoleSimt);
+    if (tensor) {
+      int rc = dipole_sub_tc(d, Q, qbar, assign_q, goff, pairs, dp.cov, dp.pw, csub, status, st);
+      if (rc != MUSE_OK) return rc;
+    } else {
+      MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_sub<T, ST, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ssub));
+      prof_mark("k_dipole_sub", st);
+      k_dipole_sub<T, ST, D><<<dim3(d.Ck, d.SB, d.B * d.Hq), 256, ssub, st>>>(d, Q, qbar, assign_q, goff, pairs, (const ST*)dp.cov,
+                                                                              (const ST*)dp.pw, csub);
+      MUSE_LAUNCH_OK();
+    }
+    round_q = tensor ? 1 : 0;
     if (sizeof(ST) == 2) {
       MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_apply<T, ST, float, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
       prof_mark("k_dipole_apply", st);
       k_dipole_apply<T, ST, float, D><<<grid, 256, smem, st>>>(d, Q, qbar, off_q, perm_q, (const float*)dp.cbar, lse_far, sel,
-                                                               (const ST*)dp.pw, dp.zall, csub, o_far, corr, zq);
+                                                               (const ST*)dp.pw, dp.zall, csub, round_q, o_far, corr, zq);
       MUSE_LAUNCH_OK();
       return MUSE_OK;
     }
@@ -444,7 +457,7 @@ static int dipole_apply_t(const Dims& d, const T* Q, const float* qbar, const in
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_apply<T, ST, ST, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prof_mark("k_dipole_apply", st);
   k_dipole_apply<T, ST, ST, D><<<grid, 256, smem, st>>>(d, Q, qbar, off_q, perm_q, (const ST*)dp.cbar, lse_far, sel, (const ST*)dp.pw,
-                                                        dp.zall, csub, o_far, corr, zq);
+                                                        dp.zall, csub, round_q, o_far, corr, zq);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }
@@ -453,14 +466,14 @@ static int dipole_apply_t(const Dims& d, const T* Q, const float* qbar, const in
 // (o_far may then be NULL).  sel, goff, pairs, csub are used with m > 0 only.
 int dipole_apply(const Dims& d, int dtype, const void* Q, const float* qbar, const int32_t* assign_q, const int32_t* off_q,
                  const int32_t* perm_q, const DipolePtrs& dp, const float* lse_far, const int32_t* sel, const int32_t* goff,
-                 const int32_t* pairs, float* csub, float* o_far, float* corr, float* zq, cudaStream_t st) {
+                 const int32_t* pairs, float* csub, float* o_far, float* corr, float* zq, int* status, cudaStream_t st) {
   typedef __nv_bfloat16 bf;
   if (dtype == MUSE_F32) {
-    if (d.D == 64) return dipole_apply_t<float, float, 64>(d, (const float*)Q, qbar, assign_q, off_q, perm_q, dp, lse_far, sel, goff, pairs, csub, o_far, corr, zq, st);
-    return dipole_apply_t<float, float, 128>(d, (const float*)Q, qbar, assign_q, off_q, perm_q, dp, lse_far, sel, goff, pairs, csub, o_far, corr, zq, st);
+    if (d.D == 64) return dipole_apply_t<float, float, 64>(d, (const float*)Q, qbar, assign_q, off_q, perm_q, dp, lse_far, sel, goff, pairs, csub, o_far, corr, zq, status, st);
+    return dipole_apply_t<float, float, 128>(d, (const float*)Q, qbar, assign_q, off_q, perm_q, dp, lse_far, sel, goff, pairs, csub, o_far, corr, zq, status, st);
   }
-  if (d.D == 64) return dipole_apply_t<bf, bf, 64>(d, (const bf*)Q, qbar, assign_q, off_q, perm_q, dp, lse_far, sel, goff, pairs, csub, o_far, corr, zq, st);
-  return dipole_apply_t<bf, bf, 128>(d, (const bf*)Q, qbar, assign_q, off_q, perm_q, dp, lse_far, sel, goff, pairs, csub, o_far, corr, zq, st);
+  if (d.D == 64) return dipole_apply_t<bf, bf, 64>(d, (const bf*)Q, qbar, assign_q, off_q, perm_q, dp, lse_far, sel, goff, pairs, csub, o_far, corr, zq, status, st);
+  return dipole_apply_t<bf, bf, 128>(d, (const bf*)Q, qbar, assign_q, off_q, perm_q, dp, lse_far, sel, goff, pairs, csub, o_far, corr, zq, status, st);
 }
 
 }  // namespace muse

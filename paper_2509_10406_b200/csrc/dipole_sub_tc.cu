@@ -1,0 +1,168 @@
+// The retrieved clusters' share of the dipole correction on the tensor cores (bf16 mode; Appendix "Error Analysis",
+// "Compatibility with Retrieval"): per (key cluster j, plane, head) group of the retrieval's inverse index
+//   out[pair][dv] = p_i(j) * sum_dk Cov_j[dv][dk] * qres[pair][dk]
+// is one GEMM [pairs x D] x [D x D].  A CTA loads the group's covariance once by TMA (K-major B operand: rows = value
+// dims), then walks the group's (query, slot) pairs in tiles of 128: the warps build the residual rows sigma (q - qbar_i)
+// as bf16 in a 128-byte-swizzled shared-memory tile (A operand), one thread issues the D / 16 tcgen05 MMAs, and every
+// thread reads its pair's row back from TMEM, scales it by the pair's centroid weight and adds it to the query's row
+// with 16-byte vector reductions.  The residuals are rounded to bf16 here, so the kernel that forms
+// (Cbar qres - this) / Z rounds them the same way (flag round_q of dipole_apply): the subtraction then still cancels
+// exactly what it should.  Every wait is bounded.
+#include <cuda.h>
+#include "common.cuh"
+#include "tc05.cuh"
+
+namespace muse {
+
+typedef __nv_bfloat16 bf16;
+int make_tmap_bf16_rows(void* out_map, const void* base, uint64_t rows, uint32_t cols, uint32_t box_rows);
+
+struct SubBars { uint64_t cov, mma; };
+
+template <int D>
+__global__ void __launch_bounds__(128)
+k_dipole_sub_tc(Dims dm, const bf16* __restrict__ Q, const float* __restrict__ qbar, const int32_t* __restrict__ assign_q,
+                const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs, const __grid_constant__ CUtensorMap tm_cov,
+                const bf16* __restrict__ pw, float* __restrict__ csub, int* __restrict__ status) {
+  constexpr int KH = D / 64;                      // 64-column halves of the K dimension
+  constexpr int TA = 128 * 128, TB = D * 128;     // bytes of one half of the A tile (128 pairs) / of the B tile (D value dims)
+  extern __shared__ __align__(1024) unsigned char sm_raw[];
+  __shared__ SubBars bars;
+  __shared__ uint32_t tbase_s;
+  __shared__ int t_s[128], i_s[128];
+  __shared__ float p_s[128];
+  unsigned char* sm = sm_raw + ((1024u - (tc::smem_u32(sm_raw) & 1023u)) & 1023u);
+  unsigned char* smA = sm;                        // [KH][128 pairs][128 B]
+  unsigned char* smB = sm + KH * TA;              // [KH][D value dims][128 B]
+  const int j = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int32_t* go = goff + (size_t)pq * (dm.SB * dm.Ck + 1) + (size_t)j * dm.SB + pl;
+  const int g0 = go[0], g1 = go[1];
+  if (g0 >= g1) return;
+  const int pk = (pq / dm.Hq) * dm.Hkv + dm.hm.g[pq % dm.Hq];
+  const int pc = dm.dipole == 2 ? pq : pk;
+  if (warp == 0) tc::tmem_alloc(&tbase_s, D);
+  if (tid == 0) {
+    tc::mbar_init(&bars.cov, 1); tc::mbar_init(&bars.mma, 1);
+    tc::mbar_init_fence();
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  tc::fence_after_sync();
+  const uint32_t tbase = tbase_s;
+  bool ok = true;
+  if (tid == 0) {
+    const int row = (((pc * dm.SB + pl) * dm.Ck) + j) * D;       // first row (value dim 0) of Cov_j
+    tc::mbar_expect_tx(&bars.cov, KH * TB);
+    for (int h = 0; h < KH; ++h) tc::tma_load_2d(smB + h * TB, &tm_cov, 64 * h, row, &bars.cov);
+  }
+  const bf16* Qp = Q + (size_t)pq * dm.N * D;
+  const int32_t* aq = assign_q + (size_t)pq * dm.N;
+  const int32_t* pr = pairs + (size_t)pq * dm.N * dm.m;
+  const bf16* pwb = pw + ((size_t)pq * dm.SB + pl) * dm.Cq * dm.Ck;
+  const uint32_t idesc = tc::idesc_bf16(128, D, 0, 0);
+  uint32_t nmma = 0;
+  for (int r0 = g0; r0 < g1; r0 += 128) {
+    {                                             // the pairs of this tile: thread = pair
+      int t = -1, i = 0;
+      if (r0 + tid < g1) {
+        t = pr[r0 + tid] / dm.m;
+        if (!MUSE_IN_RANGE(t, dm.N)) t = -1;
+      }
+      if (t >= 0) { i = aq[t]; if (!MUSE_IN_RANGE(i, dm.Cq)) { t = -1; i = 0; } }
+      t_s[tid] = t; i_s[tid] = i;
+      p_s[tid] = t >= 0 ? to_f(pwb[(size_t)i * dm.Ck + j]) : 0.f;
+    }
+    __syncthreads();
+    // residual rows as bf16 into the swizzled A tile: D / 8 lanes per row, one 16-byte chunk each
+    constexpr int LPRW = D / 8, RPI = 32 / LPRW;  // lanes per row, rows per warp iteration
+    for (int rr = warp * 32; rr < warp * 32 + 32; rr += RPI) {
+      const int r = rr + lane / LPRW, ch = lane % LPRW, t = t_s[r];
+      uint4 o = make_uint4(0u, 0u, 0u, 0u);
+      if (t >= 0) {
+        const uint4 qv = *reinterpret_cast<const uint4*>(Qp + (size_t)t * D + ch * 8);
+        const float* qb = qbar + ((size_t)pq * dm.Cq + i_s[r]) * D + ch * 8;
+        const float4 b0 = ld4(qb), b1 = ld4(qb + 4);
+        const uint32_t w[4] = {qv.x, qv.y, qv.z, qv.w};
+        const float bb[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+        uint32_t ow[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float lo = dm.sigma * (__uint_as_float(w[e] << 16) - bb[2 * e]);
+          const float hi = dm.sigma * (__uint_as_float(w[e] & 0xffff0000u) - bb[2 * e + 1]);
+          __nv_bfloat162 pk2 = __floats2bfloat162_rn(lo, hi);
+          ow[e] = *reinterpret_cast<uint32_t*>(&pk2);
+        }
+        o = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+      }
+      *reinterpret_cast<uint4*>(smA + (ch >> 3) * TA + tc::sw128_off(r, ch & 7)) = o;
+    }
+    tc::fence_async_smem();                       // the tile was written by ordinary stores and is read by the tensor core
+    __syncthreads();
+    if (tid == 0) {
+      if (nmma == 0 && !tc::mbar_wait(&bars.cov, 0)) ok = false;
+      tc::fence_after_sync();
+      if (ok) {
+        const uint32_t a0 = tc::smem_u32(smA), b0 = tc::smem_u32(smB);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks)
+          tc::mma_bf16_ss(tbase, tc::smem_desc_sw128(a0 + (ks >> 2) * TA + (ks & 3) * 32, 16, 1024),
+                          tc::smem_desc_sw128(b0 + (ks >> 2) * TB + (ks & 3) * 32, 16, 1024), idesc, ks > 0);
+      }
+      tc::mma_commit(&bars.mma);
+    }
+    __syncwarp();
+    if (!__all_sync(0xffffffffu, tc::mbar_wait(&bars.mma, nmma & 1) ? 1 : 0)) ok = false;
+    ++nmma;
+    tc::fence_after_sync();
+    const int t = t_s[tid];
+    const float p = p_s[tid];
+#pragma unroll
+    for (int q = 0; q < D / 32; ++q) {
+      float v[32];
+      tc::tmem_ld32(tbase + ((uint32_t)(warp * 32) << 16) + 32 * q, v);
+      if (ok && t >= 0) {
+        float* dst = csub + ((size_t)pq * dm.N + t) * D + 32 * q;
+#pragma unroll
+        for (int c = 0; c < 32; c += 4)
+          atomicAdd(reinterpret_cast<float4*>(dst + c), make_float4(p * v[c], p * v[c + 1], p * v[c + 2], p * v[c + 3]));
+      }
+    }
+    tc::fence_before_sync();
+    __syncthreads();                              // everyone has read the accumulator and the pair list before the next tile
+    tc::fence_after_sync();
+    if (!__syncthreads_and(ok ? 1 : 0)) { ok = false; break; }
+  }
+  tc::fence_before_sync();
+  __syncthreads();
+  if (warp == 0) tc::tmem_dealloc(tbase, D);
+  if (!ok && tid == 0) report_status(status, MUSE_STATUS_FAR_FWD_TIMEOUT);
+}
+
+bool dipole_sub_tc_supported(const Dims& d, int dtype) {
+  const long long rows = (long long)d.B * (d.dipole == 2 ? d.Hq : d.Hkv) * d.SB * d.Ck * d.D;
+  return dtype == MUSE_BF16 && rows < (1ll << 31);
+}
+
+template <int D>
+static int dipole_sub_tc_t(const Dims& d, const void* Q, const float* qbar, const int32_t* assign_q, const int32_t* goff,
+                           const int32_t* pairs, const void* cov, const void* pw, float* csub, int* status, cudaStream_t st) {
+  CUtensorMap tm;
+  const uint64_t rows = (uint64_t)d.B * (d.dipole == 2 ? d.Hq : d.Hkv) * d.SB * d.Ck * D;
+  int rc = make_tmap_bf16_rows(&tm, cov, rows, D, D);
+  if (rc != MUSE_OK) return rc;
+  const size_t smem = (size_t)(D / 64) * (128 * 128 + D * 128) + 1024;
+  MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_sub_tc<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  prof_mark("k_dipole_sub_tc", st);
+  k_dipole_sub_tc<D><<<dim3(d.Ck, d.SB, d.B * d.Hq), 128, smem, st>>>(d, (const bf16*)Q, qbar, assign_q, goff, pairs, tm, (const bf16*)pw,
+                                                                     csub, status);
+  MUSE_LAUNCH_OK();
+  return MUSE_OK;
+}
+
+int dipole_sub_tc(const Dims& d, const void* Q, const float* qbar, const int32_t* assign_q, const int32_t* goff, const int32_t* pairs,
+                  const void* cov, const void* pw, float* csub, int* status, cudaStream_t st) {
+  if (d.D == 64) return dipole_sub_tc_t<64>(d, Q, qbar, assign_q, goff, pairs, cov, pw, csub, status, st);
+  return dipole_sub_tc_t<128>(d, Q, qbar, assign_q, goff, pairs, cov, pw, csub, status, st);
+}
+
+}  // namespace muse
