@@ -93,6 +93,8 @@ def work_model(w: wl.Workload):
         # of the same contraction), and the covariance backward to the keys
         "k_dipole_sub": ("tensor", 2.0 * heads * N * m * (S - 1) / S * D * D),
         "k_dipole_bwd_pairs": ("tensor", 6.0 * heads * N * m * (S - 1) / S * D * D),
+        "k_dipole_sub_tc": ("tensor", 2.0 * heads * N * m * (S - 1) / S * D * D),
+        "k_dipole_bwd_pairs_tc": ("tensor", 4.0 * heads * N * m * (S - 1) / S * D * D),
         "k_dipole_bwd_seg": ("tensor", 4.0 * heads * N * (S - 1) / S * D * D),
         "k_dipole_dcov": ("tensor", 2.0 * heads * SB * Cq * Ck * D * D),
         "k_dipole_dpw": ("tensor", 2.0 * heads * SB * Cq * Ck * D * D),

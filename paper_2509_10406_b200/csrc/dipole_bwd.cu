@@ -602,7 +602,10 @@ static int dipole_bwd_pre_t(const Dims& d, const T* Q, const T* dO, const float*
                                                                                  dQacc, w.dcbar, w.dzs);
   }
   MUSE_LAUNCH_OK();
-  if (d.m > 0) {
+  if (d.m > 0 && sizeof(ST) == 2 && dipole_bwd_pairs_tc_supported(d, MUSE_BF16) && !path_forced(kForceDipoleSimt)) {
+    int rc = dipole_bwd_pairs_tc(d, Q, qbar, assign_q, goff, pairs, dp.cov, dp.pw, w.xq, w.dz, dQacc, w.dcov, w.dpw, status, st);
+    if (rc != MUSE_OK) return rc;
+  } else if (d.m > 0) {
     const size_t spair = (size_t)2 * (256 / (D / 4)) * kPairQ * D * sizeof(float) + (size_t)D * (D + 16 / sizeof(ST)) * sizeof(ST);
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_bwd_pairs<T, ST, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)spair));
     prof_mark("k_dipole_bwd_pairs", st);
