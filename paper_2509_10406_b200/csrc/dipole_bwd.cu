@@ -459,18 +459,32 @@ k_dipole_cov_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, co
     }
   }
   __syncthreads();
+  // a plane's dCov is fetched into registers one plane ahead, so that its latency runs under the previous plane's work
+  constexpr int NG = D * D / 4 / 256;           // float4 per thread and plane
+  float4 greg[NG];
+  auto fetch = [&](int pl) {
+    const float* g = dcov + (((size_t)pq * dm.SB + pl) * dm.Ck + j) * D * D;
+#pragma unroll
+    for (int k = 0; k < NG; ++k) {
+      const int e = tid + 256 * k;
+      greg[k] = ld4(g + (size_t)(e / (D / 4)) * D + (e % (D / 4)) * 4);
+    }
+  };
+  fetch(dm.SB - 1);
   for (int pl = dm.SB - 1; pl >= 0; --pl) {
     const float n = wb[pl];
     if (n > 0.f) {
       const float inv = 1.f / n;
-      const float* g = dcov + (((size_t)pq * dm.SB + pl) * dm.Ck + j) * D * D;
-      for (int e = tid; e < D * D / 4; e += 256) {
-        const int dv = e / (D / 4), c4 = (e % (D / 4)) * 4;
-        const float4 v = ld4(g + (size_t)dv * D + c4);
+#pragma unroll
+      for (int k = 0; k < NG; ++k) {
+        const int e = tid + 256 * k, dv = e / (D / 4), c4 = (e % (D / 4)) * 4;
         float* o = Gs + dv * (D + 1) + c4;
-        o[0] = v.x * inv; o[1] = v.y * inv; o[2] = v.z * inv; o[3] = v.w * inv;
+        o[0] = greg[k].x * inv; o[1] = greg[k].y * inv; o[2] = greg[k].z * inv; o[3] = greg[k].w * inv;
       }
       __syncthreads();
+    }
+    if (pl > 0) fetch(pl - 1);
+    if (n > 0.f) {
       for (int e = tid; e < D * D; e += 256) { const int at = (e / D) * (D + 1) + e % D; As[at] += Gs[at]; }
       if (tid < D) {
         float s = 0.f;
