@@ -276,20 +276,4 @@ size_t ret_index_elems(const Dims& d);     // int32 elements per query head
 // bsel != nullptr (k2 > 0): groups are the (cluster, chosen block) buckets, pair id = (t * m + slot) * k2 + e
 int build_ret_index(const Dims& d, const int32_t* sel, const int32_t* bsel, int32_t* scratch, RetIndex* out, cudaStream_t st);
 
-// acc[a] += sum_k M[k][d_out] * x[a][k] for NQ vectors x (rows of D floats, 16-byte aligned) against a matrix held
-// transposed in shared memory (Mt[k * (D + 1) + d_out]); the vectors are read four k at a time (one broadcast LDS.128).
-template <int D, int NQ>
-__device__ __forceinline__ void matvec_rows(const float* __restrict__ Mt, const float* __restrict__ xg, int d_out, float (&acc)[NQ]) {
-#pragma unroll 2
-  for (int k = 0; k < D; k += 4) {
-    const float c0 = Mt[(k + 0) * (D + 1) + d_out], c1 = Mt[(k + 1) * (D + 1) + d_out];
-    const float c2 = Mt[(k + 2) * (D + 1) + d_out], c3 = Mt[(k + 3) * (D + 1) + d_out];
-#pragma unroll
-    for (int a = 0; a < NQ; ++a) {
-      const float4 x = *reinterpret_cast<const float4*>(xg + a * D + k);
-      acc[a] = fmaf(c0, x.x, acc[a]); acc[a] = fmaf(c1, x.y, acc[a]); acc[a] = fmaf(c2, x.z, acc[a]); acc[a] = fmaf(c3, x.w, acc[a]);
-    }
-  }
-}
-
 }  // namespace muse

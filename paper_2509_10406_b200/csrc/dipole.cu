@@ -190,19 +190,6 @@ k_dipole_merge(Dims dm, const ST* __restrict__ P, const ST* __restrict__ cov, OT
 }
 
 // ---- 4a. the retrieved clusters' share (m > 0): one CTA per (key cluster j, plane, head) group of the inverse index ----
-constexpr int kApplyQ = 8;
-
-// Covariance (row-major [value dim][key dim]) into shared memory, transposed: Ct[key dim][value dim], pitch D + 1.
-template <class CT, int D>
-__device__ __forceinline__ void load_cov_t(const CT* __restrict__ cb, float* Ct, int tid) {
-  for (int e = tid; e < D * D / 4; e += 256) {
-    const int dv = e / (D / 4), c4 = (e % (D / 4)) * 4;
-    const float4 v = ld4(cb + (size_t)dv * D + c4);
-    Ct[(c4 + 0) * (D + 1) + dv] = v.x; Ct[(c4 + 1) * (D + 1) + dv] = v.y;
-    Ct[(c4 + 2) * (D + 1) + dv] = v.z; Ct[(c4 + 3) * (D + 1) + dv] = v.w;
-  }
-}
-
 // Register tile: a thread owns 4 consecutive value dims of kSubQ pairs; the covariance sits transposed in shared memory
 // in its storage type (Ct[key dim][value dim], rows 16-byte aligned), so that per 4 key dims a thread reads 4 vectors of
 // the matrix and kSubQ broadcast vectors of residuals for 16 * kSubQ multiply-adds -- with one value dim per thread the
@@ -294,58 +281,97 @@ k_dipole_apply(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar,
                const int32_t* __restrict__ perm_q, const CT* __restrict__ cbar, const float* __restrict__ lse_far,
                const int32_t* __restrict__ sel, const ST* __restrict__ pw, const float* __restrict__ zall,
                const float* __restrict__ csub, int round_q, float* __restrict__ o_far, float* __restrict__ corr, float* __restrict__ zq) {
-  constexpr int G = 256 / D, R = G * kApplyQ;
-  extern __shared__ float smd[];
-  float* Ct = smd;                              // [D key dims][D + 1]: transposed matrix, value dim fastest
-  float* qs = Ct + D * (D + 1);                 // [R][D] residuals
+  // same register tile as k_dipole_sub: a thread owns 4 consecutive value dims of kSubQ queries
+  constexpr int TG = D / 4, G = 256 / TG, R = G * kSubQ;
+  constexpr int P = D + 16 / (int)sizeof(CT);
+  extern __shared__ __align__(16) unsigned char smd_raw[];
+  float* qs = reinterpret_cast<float*>(smd_raw);              // [R][D] residuals
+  CT* Ct = reinterpret_cast<CT*>(qs + R * D);                 // [D key dims][P]: transposed matrix
   __shared__ float z_s[R];
+  __shared__ int t_s[R];
   const int i = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z, tid = threadIdx.x;
   const int blk = dm.causal ? pl + 1 : 0;
   const int32_t* oq = off_q + (size_t)pq * (dm.S * dm.Cq + 1) + (size_t)blk * dm.Cq + i;
   const int p0 = oq[0], p1 = oq[1];
   if (p0 >= p1) return;
-  load_cov_t<CT, D>(cbar + (((size_t)pq * dm.SB + pl) * dm.Cq + i) * D * D, Ct, tid);
+  const size_t row = ((size_t)pq * dm.SB + pl) * dm.Cq + i;
+  const CT* cb = cbar + row * D * D;
+  for (int e = tid; e < D * D; e += 256) Ct[(e % D) * P + e / D] = cb[e];          // Cbar[dv][dk] -> Ct[dk][dv]
   const float* qb = qbar + ((size_t)pq * dm.Cq + i) * D;
   const T* Qp = Q + (size_t)pq * dm.N * D;
   const int32_t* pm = perm_q + (size_t)pq * dm.N;
-  const size_t row = ((size_t)pq * dm.SB + pl) * dm.Cq + i;
-  const int grp = tid / D, dv = tid % D;
+  const int grp = tid / TG, d4 = (tid % TG) * 4;
   for (int r0 = p0; r0 < p1; r0 += R) {
     __syncthreads();
     if (tid < R) {
       float z = 1.f;
-      if (dm.m > 0 && r0 + tid < p1) {
-        const int t = pm[r0 + tid];
+      int t = -1;
+      if (r0 + tid < p1) {
+        t = pm[r0 + tid];
+        if (!MUSE_IN_RANGE(t, dm.N)) t = -1;
+      }
+      if (dm.m > 0 && t >= 0) {
         z = zall[row];
         for (int s = 0; s < dm.m; ++s) {
           const int jj = sel[((size_t)pq * dm.N + t) * dm.m + s];
           if (jj >= 0 && MUSE_IN_RANGE(jj, dm.Ck)) z -= to_f(pw[row * dm.Ck + jj]);
         }
       }
-      z_s[tid] = z;
-    }
-    for (int e = tid; e < R * D; e += 256) {
-      const int r = e / D, dk = e % D;
-      float v = r0 + r < p1 ? dm.sigma * (to_f(Qp[(size_t)pm[r0 + r] * D + dk]) - qb[dk]) : 0.f;
-      if (round_q) v = __bfloat162float(__float2bfloat16_rn(v));     // the same residuals as the tensor-core kernel that made csub
-      qs[e] = v;
+      z_s[tid] = z; t_s[tid] = t;
     }
     __syncthreads();
-    float acc[kApplyQ];
-#pragma unroll
-    for (int a = 0; a < kApplyQ; ++a) acc[a] = 0.f;
-    matvec_rows<D, kApplyQ>(Ct, qs + grp * kApplyQ * D, dv, acc);
-#pragma unroll
-    for (int a = 0; a < kApplyQ; ++a) {
-      const int r = r0 + grp * kApplyQ + a;
-      if (r < p1) {
-        const size_t t = (size_t)pq * dm.N + pm[r];
-        const float z = z_s[grp * kApplyQ + a];
-        float c = 0.f;
-        if (lse_far[t] != -INFINITY && z > 1e-30f) c = dm.m > 0 ? (acc[a] - csub[t * D + dv]) / z : acc[a];
-        if (o_far) o_far[t * D + dv] += c;
-        if (corr) { corr[t * D + dv] = c; if (dv == 0) zq[t] = z; }
+    for (int e = tid; e < R * (D / 4); e += 256) {
+      const int r = e / (D / 4), c4 = (e % (D / 4)) * 4, t = t_s[r];
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (t >= 0) {
+        const float4 q = ld4(Qp + (size_t)t * D + c4), b = ld4(qb + c4);
+        v = make_float4(dm.sigma * (q.x - b.x), dm.sigma * (q.y - b.y), dm.sigma * (q.z - b.z), dm.sigma * (q.w - b.w));
+        if (round_q) {                          // the same residuals as the tensor-core kernel that made csub
+          v.x = __bfloat162float(__float2bfloat16_rn(v.x)); v.y = __bfloat162float(__float2bfloat16_rn(v.y));
+          v.z = __bfloat162float(__float2bfloat16_rn(v.z)); v.w = __bfloat162float(__float2bfloat16_rn(v.w));
+        }
       }
+      st4(qs + r * D + c4, v);
+    }
+    __syncthreads();
+    float acc[kSubQ][4];
+#pragma unroll
+    for (int a = 0; a < kSubQ; ++a) { acc[a][0] = 0.f; acc[a][1] = 0.f; acc[a][2] = 0.f; acc[a][3] = 0.f; }
+    const float* qg = qs + grp * kSubQ * D;
+#pragma unroll 2
+    for (int dk = 0; dk < D; dk += 4) {
+      const float4 c0 = ld4(Ct + (dk + 0) * P + d4), c1 = ld4(Ct + (dk + 1) * P + d4);
+      const float4 c2 = ld4(Ct + (dk + 2) * P + d4), c3 = ld4(Ct + (dk + 3) * P + d4);
+#pragma unroll
+      for (int a = 0; a < kSubQ; ++a) {
+        const float4 q = *reinterpret_cast<const float4*>(qg + a * D + dk);
+        acc[a][0] = fmaf(c0.x, q.x, fmaf(c1.x, q.y, fmaf(c2.x, q.z, fmaf(c3.x, q.w, acc[a][0]))));
+        acc[a][1] = fmaf(c0.y, q.x, fmaf(c1.y, q.y, fmaf(c2.y, q.z, fmaf(c3.y, q.w, acc[a][1]))));
+        acc[a][2] = fmaf(c0.z, q.x, fmaf(c1.z, q.y, fmaf(c2.z, q.z, fmaf(c3.z, q.w, acc[a][2]))));
+        acc[a][3] = fmaf(c0.w, q.x, fmaf(c1.w, q.y, fmaf(c2.w, q.z, fmaf(c3.w, q.w, acc[a][3]))));
+      }
+    }
+#pragma unroll
+    for (int a = 0; a < kSubQ; ++a) {
+      const int r = grp * kSubQ + a, tl = t_s[r];
+      if (tl < 0) continue;
+      const size_t t = (size_t)pq * dm.N + tl;
+      const float z = z_s[r];
+      float4 c = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (lse_far[t] != -INFINITY && z > 1e-30f) {
+        c = make_float4(acc[a][0], acc[a][1], acc[a][2], acc[a][3]);
+        if (dm.m > 0) {
+          const float4 sb = ld4(csub + t * D + d4);
+          const float iz = 1.f / z;
+          c = make_float4((c.x - sb.x) * iz, (c.y - sb.y) * iz, (c.z - sb.z) * iz, (c.w - sb.w) * iz);
+        }
+      }
+      if (o_far) {
+        float4 o = ld4(o_far + t * D + d4);
+        o.x += c.x; o.y += c.y; o.z += c.z; o.w += c.w;
+        st4(o_far + t * D + d4, o);
+      }
+      if (corr) { st4(corr + t * D + d4, c); if (d4 == 0) zq[t] = z; }
     }
   }
 }
@@ -427,7 +453,7 @@ static int dipole_apply_t(const Dims& d, const T* Q, const float* qbar, const in
                           const int32_t* perm_q, const DipolePtrs& dp, const float* lse_far, const int32_t* sel,
                           const int32_t* goff, const int32_t* pairs, float* csub, float* o_far, float* corr, float* zq,
                           int* status, cudaStream_t st) {
-  const size_t smem = (size_t)(D * (D + 1) + (256 / D) * kApplyQ * D) * sizeof(float);
+  const size_t rows_b = (size_t)(256 / (D / 4)) * kSubQ * D * sizeof(float);      // the residual rows of one pass
   const dim3 grid(d.Cq, d.SB, d.B * d.Hq);
   int round_q = 0;
   if (d.m > 0) {
@@ -446,6 +472,7 @@ static int dipole_apply_t(const Dims& d, const T* Q, const float* qbar, const in
     }
     round_q = tensor ? 1 : 0;
     if (sizeof(ST) == 2) {
+      const size_t smem = rows_b + (size_t)D * (D + 4) * sizeof(float);
       MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_apply<T, ST, float, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
       prof_mark("k_dipole_apply", st);
       k_dipole_apply<T, ST, float, D><<<grid, 256, smem, st>>>(d, Q, qbar, off_q, perm_q, (const float*)dp.cbar, lse_far, sel,
@@ -454,6 +481,7 @@ static int dipole_apply_t(const Dims& d, const T* Q, const float* qbar, const in
       return MUSE_OK;
     }
   }
+  const size_t smem = rows_b + (size_t)D * (D + 16 / sizeof(ST)) * sizeof(ST);
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_apply<T, ST, ST, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prof_mark("k_dipole_apply", st);
   k_dipole_apply<T, ST, ST, D><<<grid, 256, smem, st>>>(d, Q, qbar, off_q, perm_q, (const ST*)dp.cbar, lse_far, sel, (const ST*)dp.pw,

@@ -27,16 +27,6 @@ namespace muse {
 
 constexpr int kDbQ = 8;                         // queries (or keys) per thread group and pass
 
-template <class CT, int D>
-__device__ __forceinline__ void db_load_t(const CT* __restrict__ cb, float* Ct, int tid, float scale) {
-  for (int e = tid; e < D * D / 4; e += 256) {
-    const int dv = e / (D / 4), c4 = (e % (D / 4)) * 4;
-    const float4 v = ld4(cb + (size_t)dv * D + c4);
-    Ct[(c4 + 0) * (D + 1) + dv] = v.x * scale; Ct[(c4 + 1) * (D + 1) + dv] = v.y * scale;
-    Ct[(c4 + 2) * (D + 1) + dv] = v.z * scale; Ct[(c4 + 3) * (D + 1) + dv] = v.w * scale;
-  }
-}
-
 // ---- per query: x_t = w_far dO / Z, delta for the far field, dZ_t -------------------------------------------------
 template <class T, int D>
 __global__ void k_dipole_bwd_prep(const T* __restrict__ dO, const float* __restrict__ LSE, const float* __restrict__ lse_far,
@@ -63,28 +53,41 @@ __global__ void k_dipole_bwd_prep(const T* __restrict__ dO, const float* __restr
 }
 
 // ---- per query segment (i, plane, head): dQ += sigma Cbar^T x,  dCbar = sum x qres^T,  sum of dZ -------------------
+// The merged matrix sits in shared memory as stored ([value dim][key dim], rows 16-byte aligned); a thread owns 4
+// consecutive key dims of kSegQ queries for Cbar^T x, and a TV x TV block of the segment's outer-product sum.
+constexpr int kSegQ = 8;
+
 template <class T, class CT, int D>
 __global__ void __launch_bounds__(256)
 k_dipole_bwd_seg(Dims dm, const T* __restrict__ Q, const float* __restrict__ qbar, const int32_t* __restrict__ off_q,
                  const int32_t* __restrict__ perm_q, const CT* __restrict__ cbar, const float* __restrict__ xq,
                  const float* __restrict__ dz, float* __restrict__ dQacc, float* __restrict__ dcbar, float* __restrict__ dzs) {
-  constexpr int G = 256 / D, R = G * kDbQ, TV = D / 16;
-  extern __shared__ float smd[];
-  float* Ct = smd;                              // Ct[dk][dv], pitch D + 1
-  float* qs = Ct + D * (D + 1);                 // [R][D] residuals
-  float* xs = qs + R * D;                       // [R][D] x rows
+  constexpr int TG = D / 4, G = 256 / TG, R = G * kSegQ, TV = D / 16;
+  constexpr int P = D + 16 / (int)sizeof(CT);
+  extern __shared__ __align__(16) unsigned char smd_raw[];
+  float* qs = reinterpret_cast<float*>(smd_raw);              // [R][D] residuals
+  float* xs = qs + R * D;                                     // [R][D] x rows
+  CT* Cs = reinterpret_cast<CT*>(xs + R * D);                 // [D value dims][P]
   __shared__ float zsum_s[R];
+  __shared__ int t_s[R];
   const int i = blockIdx.x, pl = blockIdx.y, pq = blockIdx.z, tid = threadIdx.x;
   const int blk = dm.causal ? pl + 1 : 0;
   const int32_t* oq = off_q + (size_t)pq * (dm.S * dm.Cq + 1) + (size_t)blk * dm.Cq + i;
   const int p0 = oq[0], p1 = oq[1];
   if (p0 >= p1) return;                         // dCbar and the dZ sum of an empty segment stay at their cleared zero
   const size_t row = ((size_t)pq * dm.SB + pl) * dm.Cq + i;
-  db_load_t<CT, D>(cbar + row * D * D, Ct, tid, 1.f);
+  {
+    const CT* cb = cbar + row * D * D;
+    constexpr int V = 16 / (int)sizeof(CT);
+    for (int e = tid; e < D * D / V; e += 256) {
+      const int dv = e / (D / V), c = (e % (D / V)) * V;
+      *reinterpret_cast<uint4*>(Cs + dv * P + c) = *reinterpret_cast<const uint4*>(cb + (size_t)dv * D + c);
+    }
+  }
   const float* qb = qbar + ((size_t)pq * dm.Cq + i) * D;
   const T* Qp = Q + (size_t)pq * dm.N * D;
   const int32_t* pm = perm_q + (size_t)pq * dm.N;
-  const int grp = tid / D, dk = tid % D, ty = tid >> 4, tx = tid & 15;
+  const int grp = tid / TG, d4 = (tid % TG) * 4, ty = tid >> 4, tx = tid & 15;
   float A[TV][TV];
 #pragma unroll
   for (int a = 0; a < TV; ++a)
@@ -93,34 +96,53 @@ k_dipole_bwd_seg(Dims dm, const T* __restrict__ Q, const float* __restrict__ qba
   float zacc = 0.f;
   for (int r0 = p0; r0 < p1; r0 += R) {
     __syncthreads();
-    for (int e = tid; e < R * D; e += 256) {
-      const int r = e / D, c = e % D;
-      const bool in = r0 + r < p1;
-      const size_t t = in ? (size_t)pq * dm.N + pm[r0 + r] : 0;
-      qs[e] = in ? dm.sigma * (to_f(Qp[(size_t)pm[r0 + r] * D + c]) - qb[c]) : 0.f;
-      xs[e] = in ? xq[t * D + c] : 0.f;
+    if (tid < R) {
+      int t = -1;
+      if (r0 + tid < p1) {
+        t = pm[r0 + tid];
+        if (!MUSE_IN_RANGE(t, dm.N)) t = -1;
+      }
+      t_s[tid] = t;
+      if (t >= 0) zacc += dz[(size_t)pq * dm.N + t];
     }
-    if (tid < R && r0 + tid < p1) zacc += dz[(size_t)pq * dm.N + pm[r0 + tid]];
+    __syncthreads();
+    for (int e = tid; e < R * (D / 4); e += 256) {
+      const int r = e / (D / 4), c4 = (e % (D / 4)) * 4, t = t_s[r];
+      float4 v = make_float4(0.f, 0.f, 0.f, 0.f), x = v;
+      if (t >= 0) {
+        const float4 q = ld4(Qp + (size_t)t * D + c4), b = ld4(qb + c4);
+        v = make_float4(dm.sigma * (q.x - b.x), dm.sigma * (q.y - b.y), dm.sigma * (q.z - b.z), dm.sigma * (q.w - b.w));
+        x = ld4(xq + ((size_t)pq * dm.N + t) * D + c4);
+      }
+      st4(qs + r * D + c4, v); st4(xs + r * D + c4, x);
+    }
     __syncthreads();
     // dqres[dk] = sum_dv Cbar[dv][dk] x[dv]
-    float acc[kDbQ];
+    float acc[kSegQ][4];
 #pragma unroll
-    for (int a = 0; a < kDbQ; ++a) acc[a] = 0.f;
-    // Ct is indexed [dk][dv] here and the sum runs over dv: the untransposed product, read along a row of Ct
-    const float* xg = xs + grp * kDbQ * D;
+    for (int a = 0; a < kSegQ; ++a) { acc[a][0] = 0.f; acc[a][1] = 0.f; acc[a][2] = 0.f; acc[a][3] = 0.f; }
+    const float* xg = xs + grp * kSegQ * D;
 #pragma unroll 2
     for (int dv = 0; dv < D; dv += 4) {
-      const float c0 = Ct[dk * (D + 1) + dv], c1 = Ct[dk * (D + 1) + dv + 1], c2 = Ct[dk * (D + 1) + dv + 2], c3 = Ct[dk * (D + 1) + dv + 3];
+      const float4 c0 = ld4(Cs + (dv + 0) * P + d4), c1 = ld4(Cs + (dv + 1) * P + d4);
+      const float4 c2 = ld4(Cs + (dv + 2) * P + d4), c3 = ld4(Cs + (dv + 3) * P + d4);
 #pragma unroll
-      for (int a = 0; a < kDbQ; ++a) {
+      for (int a = 0; a < kSegQ; ++a) {
         const float4 x = *reinterpret_cast<const float4*>(xg + a * D + dv);
-        acc[a] = fmaf(c0, x.x, acc[a]); acc[a] = fmaf(c1, x.y, acc[a]); acc[a] = fmaf(c2, x.z, acc[a]); acc[a] = fmaf(c3, x.w, acc[a]);
+        acc[a][0] = fmaf(c0.x, x.x, fmaf(c1.x, x.y, fmaf(c2.x, x.z, fmaf(c3.x, x.w, acc[a][0]))));
+        acc[a][1] = fmaf(c0.y, x.x, fmaf(c1.y, x.y, fmaf(c2.y, x.z, fmaf(c3.y, x.w, acc[a][1]))));
+        acc[a][2] = fmaf(c0.z, x.x, fmaf(c1.z, x.y, fmaf(c2.z, x.z, fmaf(c3.z, x.w, acc[a][2]))));
+        acc[a][3] = fmaf(c0.w, x.x, fmaf(c1.w, x.y, fmaf(c2.w, x.z, fmaf(c3.w, x.w, acc[a][3]))));
       }
     }
 #pragma unroll
-    for (int a = 0; a < kDbQ; ++a) {
-      const int r = r0 + grp * kDbQ + a;
-      if (r < p1) dQacc[((size_t)pq * dm.N + pm[r]) * D + dk] += dm.sigma * acc[a];
+    for (int a = 0; a < kSegQ; ++a) {
+      const int t = t_s[grp * kSegQ + a];
+      if (t < 0) continue;
+      float* dst = dQacc + ((size_t)pq * dm.N + t) * D + d4;      // this segment owns the query: plain read-modify-write
+      float4 o = ld4(dst);
+      o.x += dm.sigma * acc[a][0]; o.y += dm.sigma * acc[a][1]; o.z += dm.sigma * acc[a][2]; o.w += dm.sigma * acc[a][3];
+      st4(dst, o);
     }
     // dCbar[dv][dk] += x[dv] qres[dk]; thread (ty, tx) owns value dims ty*TV.., key dims tx*TV..
     for (int r = 0; r < R; ++r) {
@@ -603,8 +625,9 @@ static int dipole_bwd_pre_t(const Dims& d, const T* Q, const T* dO, const float*
   MUSE_CUDA_OK(cudaMemsetAsync(w.dcbar, 0, segs * D * D * sizeof(float), st));
   MUSE_CUDA_OK(cudaMemsetAsync(w.dzs, 0, segs * sizeof(float), st));
   MUSE_CUDA_OK(cudaMemsetAsync(w.dpw, 0, segs * d.Ck * sizeof(float), st));
-  const size_t smem = (size_t)(D * (D + 1) + 2 * (256 / D) * kDbQ * D) * sizeof(float);
+  const size_t rows_b = (size_t)2 * (256 / (D / 4)) * kSegQ * D * sizeof(float);
   const bool f32bar = d.m > 0 || sizeof(ST) == 4;
+  const size_t smem = rows_b + (f32bar ? (size_t)D * (D + 4) * sizeof(float) : (size_t)D * (D + 16 / sizeof(ST)) * sizeof(ST));
   prof_mark("k_dipole_bwd_seg", st);
   if (f32bar) {
     MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_bwd_seg<T, float, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
