@@ -231,3 +231,29 @@ def test_tilted_dipole_forward_and_backward_match_oracle(name):
             assert rel_err(got, e) < rel_err(got, plain), key
     if w.dtype == "f32":
         assert far_apart > 4 * t and max(moved.values()) > 4 * t
+
+
+@pytest.mark.parametrize("dipole", [1, 2])
+def test_dipole_backward_rebuilds_summaries_when_not_given(dipole):
+    """muse_attn_bwd with summaries == NULL rebuilds them (with the dipole's arrays and, for dipole == 2, the tilt point)
+    in the tail of its scratch: same gradients as with the forward's buffer."""
+    from paper_2509_10406_b200 import binding as mb
+    w = CASES["tiny"].with_(m=2)
+    c = Case(w, gain=128.0)
+    qbar32 = c.qbar.astype(np.float32)
+    p = c.params(dipole=dipole)
+    buf = mb.MuseBuffers(p, backward=True)
+    Q, K, V, dO = c.dev()
+    aq, qb = to_dev(c.a_q, "i"), to_dev(qbar32, "f32")
+    if dipole == 2:
+        mb.muse_dipole_tilt_point(p, aq, qb, buf.summaries)
+    mb.muse_summarize(p, K, V, to_dev(c.a_k, "i"), qb, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
+    mb.muse_attn_fwd(p, Q, K, V, aq, qb, buf.off_k, buf.perm_k, buf.summaries, None, buf.O, buf.LSE, buf.sel, buf.ws)
+    res = []
+    for summ, ws in ((buf.summaries, buf.ws), (None, torch.empty(buf.sizes[5], dtype=torch.uint8, device="cuda"))):
+        mb.muse_attn_bwd(p, Q, K, V, buf.O, buf.LSE, dO, aq, qb, buf.off_k, buf.perm_k, summ, buf.sel, buf.dQ, buf.dK, buf.dV, ws)
+        torch.cuda.synchronize()
+        assert mb.muse_status(ws) == 0
+        res.append((to_np(buf.dQ).copy(), to_np(buf.dK).copy(), to_np(buf.dV).copy()))
+    for a, b in zip(*res):
+        assert rel_err(b, a) <= 1e-5
