@@ -213,9 +213,9 @@ bool dipole_bwd_tc_supported(const Dims& d, int dtype);
 bool dipole_bwd_pairs_tc_supported(const Dims& d, int dtype);
 int dipole_bwd_pairs_tc(const Dims& d, const void* Q, const float* qbar, const int32_t* assign_q, const int32_t* goff,
                         const int32_t* pairs, const void* cov, const void* pw, const float* xq, const float* dz, float* dQacc,
-                        float* dcov, float* dpw, int* status, cudaStream_t st);
+                        float* dcov, float* dpw, int fill_empty, int* status, cudaStream_t st);
 int dipole_bwd_tc(const Dims& d, const void* P, const void* cov, const float* dcbar, void* dcbar_bf, const float* dzs, float* dcov,
-                  float* dpw, int with_dpw, int dcov_has_terms, int* status, cudaStream_t st);
+                  float* dpw, int with_dpw, const int32_t* goff, int* status, cudaStream_t st);
 int dipole_tilt_point(const Dims& d, const int32_t* assign_q, const float* qbar, float* qstar, cudaStream_t st);
 int far_fwd_again(const Dims& d, int dtype, const void* Q, const float* qbar, const int32_t* off_q, const int32_t* perm_q,
                   const SummPtrs& sp, const int32_t* sel_in, int32_t* sel_tmp, float* o_far, float* lse_far, int* status,

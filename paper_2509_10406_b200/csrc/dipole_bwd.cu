@@ -639,8 +639,10 @@ static int dipole_bwd_pre_t(const Dims& d, const T* Q, const T* dO, const float*
                                                                                  dQacc, w.dcbar, w.dzs);
   }
   MUSE_LAUNCH_OK();
+  const bool tensor = dipole_bwd_tc_supported(d, sizeof(ST) == 2 ? MUSE_BF16 : MUSE_F32) && !path_forced(kForceDipoleSimt);
   if (d.m > 0 && sizeof(ST) == 2 && dipole_bwd_pairs_tc_supported(d, MUSE_BF16) && !path_forced(kForceDipoleSimt)) {
-    int rc = dipole_bwd_pairs_tc(d, Q, qbar, assign_q, goff, pairs, dp.cov, dp.pw, w.xq, w.dz, dQacc, w.dcov, w.dpw, status, st);
+    int rc = dipole_bwd_pairs_tc(d, Q, qbar, assign_q, goff, pairs, dp.cov, dp.pw, w.xq, w.dz, dQacc, w.dcov, w.dpw, tensor ? 0 : 1,
+                                 status, st);
     if (rc != MUSE_OK) return rc;
   } else if (d.m > 0) {
     const size_t spair = (size_t)2 * (256 / (D / 4)) * kPairQ * D * sizeof(float) + (size_t)D * (D + 16 / sizeof(ST)) * sizeof(ST);
@@ -650,12 +652,11 @@ static int dipole_bwd_pre_t(const Dims& d, const T* Q, const T* dO, const float*
                                                                                    (const ST*)dp.pw, w.xq, w.dz, dQacc, w.dcov, w.dpw);
     MUSE_LAUNCH_OK();
   }
-  const bool tensor = dipole_bwd_tc_supported(d, sizeof(ST) == 2 ? MUSE_BF16 : MUSE_F32) && !path_forced(kForceDipoleSimt);
   if (d.m == 0 && !tensor) {                              // the plain kernel adds to dCov; the tensor kernel can overwrite it
     prof_mark("memset", st);
     MUSE_CUDA_OK(cudaMemsetAsync(w.dcov, 0, pq * d.SB * d.Ck * D * D * sizeof(float), st));
   }
-  if (tensor) return dipole_bwd_tc(d, dp.pw, dp.cov, w.dcbar, w.dcbar_bf, w.dzs, w.dcov, w.dpw, d.agg_grad, d.m > 0 ? 1 : 0, status, st);
+  if (tensor) return dipole_bwd_tc(d, dp.pw, dp.cov, w.dcbar, w.dcbar_bf, w.dzs, w.dcov, w.dpw, d.agg_grad, d.m > 0 ? goff : nullptr, status, st);
   prof_mark("k_dipole_dcov", st);
   k_dipole_dcov<ST><<<dim3(D * D / 256, cdiv(d.Ck, kDcJ), (unsigned)(pq * d.SB)), 256, 0, st>>>(d, (const ST*)dp.pw, w.dcbar, w.dcov);
   MUSE_LAUNCH_OK();

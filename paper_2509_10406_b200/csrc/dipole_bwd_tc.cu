@@ -35,7 +35,8 @@ __global__ void k_to_bf16(const float* __restrict__ src, size_t n4, bf16* __rest
 template <int MODE>
 __global__ void __launch_bounds__(128)
 k_dipole_bwd_gemm_tc(Dims dm, const __grid_constant__ CUtensorMap tm_a, const __grid_constant__ CUtensorMap tm_b,
-                     const float* __restrict__ dzs, float* __restrict__ out, int accumulate, int* __restrict__ status) {
+                     const float* __restrict__ dzs, float* __restrict__ out, int accumulate, const int32_t* __restrict__ goff,
+                     int* __restrict__ status) {
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ DbBars bars;
   __shared__ uint32_t tbase_s;
@@ -111,6 +112,11 @@ k_dipole_bwd_gemm_tc(Dims dm, const __grid_constant__ CUtensorMap tm_a, const __
   const int rows = MODE == 0 ? dm.Ck : dm.Cq, cols = MODE == 0 ? DD : dm.Ck;
   float* orow = out + ((size_t)pp * rows + r) * cols + n0;
   const float add = MODE == 1 && r < rows ? dzs[(size_t)pp * dm.Cq + r] : 0.f;
+  if (MODE == 0 && goff != nullptr && r < rows) {
+    // dCov rows of clusters that no query retrieved in this plane were left unwritten by the per-pair kernel: overwrite
+    const int32_t* go = goff + (size_t)pq * (dm.SB * dm.Ck + 1) + (size_t)r * dm.SB + pl;
+    accumulate = go[1] > go[0] ? 1 : 0;
+  }
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     float v[32];
@@ -144,9 +150,10 @@ bool dipole_bwd_tc_supported(const Dims& d, int dtype) {
 }
 
 // dcbar_bf: scratch for the bf16 copy of dCbar ([B*Hq*SB*Cq][D*D]).
-// dcov_has_terms: dCov already holds the retrieved clusters' (negative) share and is added to; otherwise it is overwritten.
+// goff != NULL (m > 0): the rows of dCov whose (cluster, plane) group of the inverse index has pairs already hold the retrieved
+// clusters' (negative) share and are added to; every other row is overwritten.
 int dipole_bwd_tc(const Dims& d, const void* P, const void* cov, const float* dcbar, void* dcbar_bf, const float* dzs, float* dcov,
-                  float* dpw, int with_dpw, int dcov_has_terms, int* status, cudaStream_t st) {
+                  float* dpw, int with_dpw, const int32_t* goff, int* status, cudaStream_t st) {
   const int DD = d.D * d.D;
   const uint64_t rows_p = (uint64_t)d.B * d.Hq * d.SB * d.Cq, rows_c = (uint64_t)d.B * (d.dipole == 2 ? d.Hq : d.Hkv) * d.SB * d.Ck;
   const size_t n4 = rows_p * DD / 4;
@@ -163,11 +170,11 @@ int dipole_bwd_tc(const Dims& d, const void* P, const void* cov, const float* dc
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_bwd_gemm_tc<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_bwd_gemm_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prof_mark("k_dipole_dcov_tc", st);
-  k_dipole_bwd_gemm_tc<0><<<dim3(DD / 128, cdiv(d.Ck, 128), d.B * d.Hq * d.SB), 128, smem, st>>>(d, tp64, tg64, nullptr, dcov, dcov_has_terms, status);
+  k_dipole_bwd_gemm_tc<0><<<dim3(DD / 128, cdiv(d.Ck, 128), d.B * d.Hq * d.SB), 128, smem, st>>>(d, tp64, tg64, nullptr, dcov, 0, goff, status);
   MUSE_LAUNCH_OK();
   if (with_dpw) {
     prof_mark("k_dipole_dpw_tc", st);
-    k_dipole_bwd_gemm_tc<1><<<dim3(cdiv(d.Ck, 128), cdiv(d.Cq, 128), d.B * d.Hq * d.SB), 128, smem, st>>>(d, tg128, tc128, dzs, dpw, 1, status);
+    k_dipole_bwd_gemm_tc<1><<<dim3(cdiv(d.Ck, 128), cdiv(d.Cq, 128), d.B * d.Hq * d.SB), 128, smem, st>>>(d, tg128, tc128, dzs, dpw, 1, nullptr, status);
     MUSE_LAUNCH_OK();
   }
   return MUSE_OK;

@@ -150,7 +150,8 @@ __global__ void __launch_bounds__(128)
 k_dipole_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const float* __restrict__ qbar, const int32_t* __restrict__ assign_q,
                       const int32_t* __restrict__ goff, const int32_t* __restrict__ pairs, const __grid_constant__ CUtensorMap tm_cov,
                       const bf16* __restrict__ pw, const float* __restrict__ xq, const float* __restrict__ dz,
-                      float* __restrict__ dQacc, float* __restrict__ dcov, float* __restrict__ dpw, int* __restrict__ status) {
+                      float* __restrict__ dQacc, float* __restrict__ dcov, float* __restrict__ dpw, int fill_empty,
+                      int* __restrict__ status) {
   constexpr int D = 128, TA = 128 * 128;          // one 64-column half of a [128 rows][D] bf16 tile
   extern __shared__ __align__(1024) unsigned char sm_raw[];
   __shared__ PairBars bars;
@@ -167,7 +168,8 @@ k_dipole_bwd_pairs_tc(Dims dm, const bf16* __restrict__ Q, const float* __restri
   const int g0 = go[0], g1 = go[1];
   float* out = dcov + (((size_t)pq * dm.SB + pl) * dm.Ck + j) * D * D;
   if (g0 >= g1) {                                 // no pair retrieved this cluster in this plane: its share is zero
-    for (int e = tid; e < D * D / 4; e += 128) reinterpret_cast<float4*>(out)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (fill_empty)                               // (the tensor-core contraction that follows overwrites such rows itself)
+      for (int e = tid; e < D * D / 4; e += 128) reinterpret_cast<float4*>(out)[e] = make_float4(0.f, 0.f, 0.f, 0.f);
     return;
   }
   const int pk = (pq / dm.Hq) * dm.Hkv + dm.hm.g[pq % dm.Hq];
@@ -308,7 +310,7 @@ bool dipole_bwd_pairs_tc_supported(const Dims& d, int dtype) {
 
 int dipole_bwd_pairs_tc(const Dims& d, const void* Q, const float* qbar, const int32_t* assign_q, const int32_t* goff,
                         const int32_t* pairs, const void* cov, const void* pw, const float* xq, const float* dz, float* dQacc,
-                        float* dcov, float* dpw, int* status, cudaStream_t st) {
+                        float* dcov, float* dpw, int fill_empty, int* status, cudaStream_t st) {
   CUtensorMap tm;
   const uint64_t rows = (uint64_t)d.B * (d.dipole == 2 ? d.Hq : d.Hkv) * d.SB * d.Ck * d.D;
   int rc = make_tmap_bf16_rows(&tm, cov, rows, d.D, d.D);
@@ -317,7 +319,7 @@ int dipole_bwd_pairs_tc(const Dims& d, const void* Q, const float* qbar, const i
   MUSE_CUDA_OK(cudaFuncSetAttribute(k_dipole_bwd_pairs_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   prof_mark("k_dipole_bwd_pairs_tc", st);
   k_dipole_bwd_pairs_tc<<<dim3(d.Ck, d.SB, d.B * d.Hq), 128, smem, st>>>(d, (const bf16*)Q, qbar, assign_q, goff, pairs, tm, (const bf16*)pw,
-                                                                        xq, dz, dQacc, dcov, dpw, status);
+                                                                        xq, dz, dQacc, dcov, dpw, fill_empty, status);
   MUSE_LAUNCH_OK();
   return MUSE_OK;
 }
