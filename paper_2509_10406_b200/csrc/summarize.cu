@@ -261,7 +261,7 @@ static int summarize_t(const Dims& d, int dtype, const T* K, const T* V, const i
   void* qsplit = ar.take<__nv_bfloat16>(2 * (size_t)d.B * d.Hq * d.Cq * d.D);   // split centroids for the tensor kernel
   rc = summarize_planes<T, D>(d, dtype, Kp, Vp, off_k, qbar, summ_ptrs(L, base), 0, qsplit, status, st);
   if (rc == MUSE_OK && d.k2 > 0) rc = summarize_planes<T, D>(d, dtype, Kp, Vp, off_k, qbar, summ_ptrs_blk(L, base), 1, qsplit, status, st);
-  if (rc != MUSE_OK || !d.dipole) return rc;
+  if (rc != MUSE_OK || !d.dipole || d.SB == 0) return rc;     // one causal block: no far field, nothing to correct
   return dipole_build(d, dtype, Kp, Vp, off_k, summ_ptrs(L, base).mu, dipole_ptrs(L, base), status, st);
 }
 

@@ -257,3 +257,43 @@ def test_dipole_backward_rebuilds_summaries_when_not_given(dipole):
         res.append((to_np(buf.dQ).copy(), to_np(buf.dK).copy(), to_np(buf.dV).copy()))
     for a, b in zip(*res):
         assert rel_err(b, a) <= 1e-5
+
+
+def test_dipole_with_selection_per_query_cluster_and_with_a_single_block():
+    """Selection per query cluster (every query of a segment retrieves the same clusters) next to the dipole, forward and
+    backward; and one causal block (no far field at all): the dipole then changes nothing and nothing faults."""
+    from paper_2509_10406_b200 import binding as mb
+    w = CASES["tiny"].with_(m=2)
+    c = Case(w, gain=128.0)
+    qbar32 = c.qbar.astype(np.float32)
+    Q, K, V, dO = c.dev()
+    aq, qb = to_dev(c.a_q, "i"), to_dev(qbar32, "f32")
+    args = (c.Q.astype(np.float64), c.K.astype(np.float64), c.V.astype(np.float64), c.dO.astype(np.float64), c.a_q, c.a_k,
+            qbar32.astype(np.float64))
+
+    def run(p):
+        buf = mb.MuseBuffers(p, backward=True)
+        if p.dipole == 2:
+            mb.muse_dipole_tilt_point(p, aq, qb, buf.summaries)
+        mb.muse_summarize(p, K, V, to_dev(c.a_k, "i"), qb, buf.off_k, buf.perm_k, buf.summaries, buf.ws)
+        mb.muse_attn_fwd(p, Q, K, V, aq, qb, buf.off_k, buf.perm_k, buf.summaries, None, buf.O, buf.LSE, buf.sel, buf.ws)
+        mb.muse_attn_bwd(p, Q, K, V, buf.O, buf.LSE, dO, aq, qb, buf.off_k, buf.perm_k, buf.summaries, buf.sel, buf.dQ, buf.dK, buf.dV, buf.ws)
+        torch.cuda.synchronize()
+        assert mb.muse_status(buf.ws) == 0
+        return to_np(buf.O), to_np(buf.dQ), to_np(buf.dK), to_np(buf.dV), to_np(buf.sel)[..., :w.m]
+
+    O, dQ, dK, dV, sel = run(c.params(dipole=2, sel_mode=1))
+    kw = dict(sigma=c.sigma, S=w.S, Ck=w.Ck, m=w.m, sel=sel, sel_mode=1, dipole=2)
+    eO, _, _ = orc.layer_forward(*args[:3], *args[4:], **kw)
+    eQ, eK, eV = orc.layer_backward(*args, **kw)
+    for got, ref in ((O, eO), (dQ, eQ), (dK, eK), (dV, eV)):
+        assert rel_err(got, ref) <= 1e-4
+    # every query of a segment carries its cluster's selection
+    Bs = w.N // w.S
+    for t in range(Bs, w.N, 37):
+        same = (c.a_q[0, 0] == c.a_q[0, 0, t]) & (np.arange(w.N) // Bs == t // Bs)
+        assert (sel[0, 0][same] == sel[0, 0, t]).all()
+    one = run(c.params(dipole=1, n_blocks=1))
+    ref = run(c.params(dipole=0, n_blocks=1))
+    for a, b in zip(one[:4], ref[:4]):
+        np.testing.assert_array_equal(a, b)
