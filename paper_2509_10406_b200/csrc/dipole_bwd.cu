@@ -412,8 +412,8 @@ k_dipole_cov_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, co
                  float* __restrict__ dK_perm, float* __restrict__ dV_perm) {
   extern __shared__ float smd[];
   float* As = smd;                              // As[dv][dk], pitch D + 1: sum over later planes of dCov / n
-  float* Gs = As + D * (D + 1);                 // this plane's dCov / n
-  float* kb = Gs + D * (D + 1);                 // [SB][D] prefix means of k - k0
+  float* avp = As + D * (D + 1);                // [8 warps][D] partial column sums of a plane
+  float* kb = avp + 8 * D;                      // [SB][D] prefix means of k - k0
   float* vb = kb + dm.SB * D;                   // [SB][D] prefix means of v
   float* ks = vb + dm.SB * D;                   // [kDbQ][D]
   float* vs = ks + kDbQ * D;
@@ -496,39 +496,49 @@ k_dipole_cov_bwd(Dims dm, const T* __restrict__ Kp, const T* __restrict__ Vp, co
   for (int pl = dm.SB - 1; pl >= 0; --pl) {
     const float n = wb[pl];
     if (n > 0.f) {
+      // straight from the registers: A += G / n (every thread its own elements); row sums against km (the D / 4 lanes
+      // that share a row reduce by shuffles) and column sums against vm (per-warp partials, then one pass over the warps)
       const float inv = 1.f / n;
+      const ST* cv = cov + (((size_t)pq * dm.SB + pl) * dm.Ck + j) * D * D;
+      float av4[4] = {0.f, 0.f, 0.f, 0.f}, cc = 0.f;
 #pragma unroll
       for (int k = 0; k < NG; ++k) {
         const int e = tid + 256 * k, dv = e / (D / 4), c4 = (e % (D / 4)) * 4;
-        float* o = Gs + dv * (D + 1) + c4;
-        o[0] = greg[k].x * inv; o[1] = greg[k].y * inv; o[2] = greg[k].z * inv; o[3] = greg[k].w * inv;
+        const float4 g = make_float4(greg[k].x * inv, greg[k].y * inv, greg[k].z * inv, greg[k].w * inv);
+        float* o = As + dv * (D + 1) + c4;
+        o[0] += g.x; o[1] += g.y; o[2] += g.z; o[3] += g.w;
+        const float* kp = kb + pl * D + c4;
+        float part = g.x * kp[0] + g.y * kp[1] + g.z * kp[2] + g.w * kp[3];
+#pragma unroll
+        for (int o2 = D / 8; o2 > 0; o2 >>= 1) part += __shfl_xor_sync(0xffffffffu, part, o2);
+        const float vm = vb[pl * D + dv];
+        if (lane % (D / 4) == 0) {
+          ak[dv] += part;
+          if (TILT && dm.agg_grad) cc = fmaf(part, vm, cc);          // vm^T (dCov / W) km
+        }
+        av4[0] = fmaf(g.x, vm, av4[0]); av4[1] = fmaf(g.y, vm, av4[1]); av4[2] = fmaf(g.z, vm, av4[2]); av4[3] = fmaf(g.w, vm, av4[3]);
+        if (TILT && dm.agg_grad) {              // - <dCov / W, Cov> with the stored covariance
+          const float4 c = ld4(cv + (size_t)dv * D + c4);
+          cc -= g.x * c.x + g.y * c.y + g.z * c.z + g.w * c.w;
+        }
       }
-      __syncthreads();
+      if (D == 64) {                            // two rows per warp pass: the half-warps hold the same columns
+#pragma unroll
+        for (int i = 0; i < 4; ++i) av4[i] += __shfl_xor_sync(0xffffffffu, av4[i], 16);
+      }
+      if (lane < D / 4) { float* o = avp + warp * D + lane * 4; o[0] = av4[0]; o[1] = av4[1]; o[2] = av4[2]; o[3] = av4[3]; }
+      if (TILT && dm.agg_grad) {
+        cc = warp_sum(cc);
+        if (lane == 0) atomicAdd(&s_suf, cc);
+      }
     }
     if (pl > 0) fetch(pl - 1);
-    if (n > 0.f) {
-      for (int e = tid; e < D * D; e += 256) { const int at = (e / D) * (D + 1) + e % D; As[at] += Gs[at]; }
-      if (tid < D) {
-        float s = 0.f;
-        for (int dk = 0; dk < D; ++dk) s = fmaf(Gs[tid * (D + 1) + dk], kb[pl * D + dk], s);
-        ak[tid] += s;
-        if (TILT && dm.agg_grad) {              // vm^T (dCov / W) km, over the D value dims
-          const float part = warp_sum(s * vb[pl * D + tid]);
-          if (lane == 0) atomicAdd(&s_suf, part);
-        }
-      } else if (tid < 2 * D) {
-        const int dk = tid - D;
-        float s = 0.f;
-        for (int dv = 0; dv < D; ++dv) s = fmaf(Gs[dv * (D + 1) + dk], vb[pl * D + dv], s);
-        av[dk] += s;
-      }
-      if (TILT && dm.agg_grad) {                // - <dCov / W, Cov> with the stored covariance
-        const ST* cv = cov + (((size_t)pq * dm.SB + pl) * dm.Ck + j) * D * D;
-        float part = 0.f;
-        for (int e = tid; e < D * D; e += 256) part = fmaf(Gs[(e / D) * (D + 1) + e % D], to_f(cv[e]), part);
-        part = warp_sum(part);
-        if (lane == 0) atomicAdd(&s_suf, -part);
-      }
+    __syncthreads();
+    if (n > 0.f && tid < D) {
+      float s = 0.f;
+#pragma unroll
+      for (int w2 = 0; w2 < 8; ++w2) s += avp[w2 * D + tid];
+      av[tid] += s;
     }
     __syncthreads();
     // keys of bucket (j, block pl): every plane >= pl holds them
@@ -605,7 +615,7 @@ DipoleBwdWs dipole_bwd_ws(const Dims& d, Arena& ar) {
 }
 
 bool dipole_bwd_supported(const Dims& d) {
-  const size_t smem = (size_t)(2 * d.D * (d.D + 1) + 2 * d.SB * d.D + 2 * kDbQ * d.D + 4 * d.D + d.SB) * sizeof(float);
+  const size_t smem = (size_t)(d.D * (d.D + 1) + 8 * d.D + 2 * d.SB * d.D + 2 * kDbQ * d.D + 4 * d.D + d.SB) * sizeof(float);
   return smem <= 200 * 1024;
 }
 
@@ -693,7 +703,7 @@ int dipole_bwd_dmu(const Dims& d, int dtype, const DipolePtrs& dp, const DipoleB
 template <class T, class ST, int D>
 static int dipole_bwd_keys_t(const Dims& d, const T* Kp, const T* Vp, const int32_t* off_k, const DipolePtrs& dp, const DipoleBwdWs& w,
                              float* dK_perm, float* dV_perm, cudaStream_t st) {
-  const size_t smem = (size_t)(2 * D * (D + 1) + 2 * d.SB * D + 2 * kDbQ * D + 4 * D + d.SB) * sizeof(float);
+  const size_t smem = (size_t)(D * (D + 1) + 8 * D + 2 * d.SB * D + 2 * kDbQ * D + 4 * D + d.SB) * sizeof(float);
   const dim3 grid(d.Ck, d.B * d.Hq);
   prof_mark("k_dipole_cov_bwd", st);
   if (d.dipole == 2) {
