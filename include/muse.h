@@ -317,8 +317,8 @@ MUSE_API long muse_profile_report(char* buf, size_t cap);
  * muse_test_force_paths: bit mask; a set bit makes later calls take the library's other kernel
  *   for one step at shapes where the tensor-core kernel is the default (1 summaries, 2 far field
  *   forward and backward, 4 key-side summary backward, 8 retrieval forward per (cluster, plane)
- *   group, 16 retrieval backward as separate dQ and dK/dV kernels, 32 dipole merge and the two dense
- *   contractions of the dipole's backward, 64 block
+ *   group, 16 retrieval backward as separate dQ and dK/dV kernels, 32 every tensor-core kernel of the
+ *   dipole correction (merge, per-pair products, the dense contractions of its backward), 64 block
  *   selection of the two-level retrieval with a warp per query); 0 restores the default.
  *   Process-wide.
  * muse_test_wait_timeout: clears the status words of `ws` (>= 256 bytes) and launches a one-warp
